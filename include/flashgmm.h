@@ -1,0 +1,130 @@
+/* flashgmm.h -- C ABI of libflashgmm: fused EM iteration of a diagonal-covariance Gaussian mixture on one
+ * NVIDIA B200 (sm_100a).
+ *
+ * Model (paper Section 2, generalised from sigma_k^2 I to a per-dimension variance):
+ *     p(x) = sum_k pi_k N(x | mu_k, diag(var_k)),   log z_ik = log pi_k + log N(x_i | mu_k, diag(var_k)),
+ *     r_ik = z_ik / sum_j z_ij  (evaluated in log space with a log-sum-exp shift).
+ * One EM iteration (paper Eq. 1-3 and Algorithm 1) is computed without ever storing the N x K responsibility
+ * matrix: only the sufficient statistics
+ *     N_k = sum_i r_ik,   S1_kd = sum_i r_ik x_id,   S2_kd = sum_i r_ik x_id^2,   loglik = sum_i log sum_k z_ik
+ * leave the chip (Algorithm 1's M_k is S1; its scalar Q_k is replaced by S2 so that the variance can use the NEW
+ * mean as Eq. 3 requires).  Device memory used beyond the caller's arrays is gmm_scratch_bytes(D, K): it does not
+ * grow with N (paper Section 3.2, "Peak memory use").
+ *
+ * Conventions
+ *   - "device" pointers are CUDA device pointers on the context's device; "host" pointers are ordinary host memory.
+ *   - Layout: X is row-major [N x D] float32; mu, var, S1, S2 are row-major [K x D]; pi, Nk are [K].
+ *   - Ownership: the caller owns every array it passes.  The library owns only the context's scratch, which it
+ *     allocates at gmm_create / first use of a larger (D, K) and frees in gmm_destroy.
+ *   - Every function returns GMM_OK (0) or a negative error code and never throws or aborts.  After a failure
+ *     gmm_last_error(ctx) gives a human-readable message.  Output arrays are unspecified after a failure.
+ *   - Work is enqueued on the context's stream; a call that has a host output synchronises that stream before it
+ *     returns, calls without host outputs (gmm_finalize, gmm_assign_topm) return with the work still in flight.
+ *   - Results are deterministic: the same inputs give the same bits on every call (no floating-point atomics;
+ *     per-CTA partial sums are added in a fixed order in float64).
+ *   - A context is not thread-safe; use one per host thread.
+ */
+#ifndef FLASHGMM_H
+#define FLASHGMM_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define GMM_OK        0
+#define GMM_EINVAL   -1   /* null pointer, N/D/K/m/iters out of range, negative floor */
+#define GMM_EALIGN   -2   /* a pointer is not aligned for its element type */
+#define GMM_ENOMEM   -3   /* scratch allocation failed */
+#define GMM_ECUDA    -4   /* a CUDA call failed; message in gmm_last_error */
+#define GMM_ENUMERIC -5   /* var <= 0, pi < 0, non-finite parameter, or non-finite log-likelihood */
+#define GMM_ETIMEOUT -6   /* a bounded device-side wait expired; results invalid */
+#define GMM_EUNSUPPORTED -7 /* the requested kernel path cannot run this shape */
+
+/* Kernel paths (gmm_set_path).  AUTO picks the tensor-core path when the shape allows it. */
+#define GMM_PATH_AUTO   0
+#define GMM_PATH_FP32   1  /* CUDA-core float32 kernels with direct differences (x - mu)^2 / var; any shape */
+#define GMM_PATH_TENSOR 2  /* tcgen05 tensor-core kernels on the expanded quadratic form; restricted shapes */
+
+#define GMM_MAX_TOPM 8
+
+typedef struct gmm_ctx gmm_ctx;
+
+/* Create a context on CUDA device `device`.  `cuda_stream` is a cudaStream_t (NULL = the legacy default stream) on
+ * which all work of this context is enqueued; the caller keeps ownership of the stream. */
+int gmm_create(gmm_ctx** out, int device, void* cuda_stream);
+int gmm_destroy(gmm_ctx* ctx);
+
+/* Select the kernel path for later calls (default GMM_PATH_AUTO).  GMM_EUNSUPPORTED is reported by the compute
+ * call, not here, if a forced path cannot run the shape. */
+int gmm_set_path(gmm_ctx* ctx, int path);
+/* The path (GMM_PATH_FP32 or GMM_PATH_TENSOR) the most recent compute call actually ran. */
+int gmm_last_path(const gmm_ctx* ctx);
+
+/* E-step and sufficient statistics under the INPUT parameters (paper Section 2 responsibilities; Eq. 1; the
+ * numerators of Eq. 2 and Eq. 3; Algorithm 1 without its last line).
+ *   X [N x D] device; pi [K], mu [K x D], var [K x D] device float32, var > 0, pi >= 0.
+ *   Nk [K], S1 [K x D], S2 [K x D] device float64 outputs (overwritten).
+ *   loglik: host output, total log-likelihood sum_i log sum_k z_ik under the input parameters (natural log,
+ *           including the -(D/2) log(2 pi) constant).
+ * Synchronises the stream.  1 <= N, 1 <= D, 1 <= K. */
+int gmm_em_step(gmm_ctx* ctx, const float* X, int64_t N, int D, int K,
+                const float* pi, const float* mu, const float* var,
+                double* Nk, double* S1, double* S2, double* loglik);
+
+/* The same statistics with X in HOST memory (pageable or pinned): the library streams X through two device
+ * staging buffers, overlapping the copy of one chunk with the kernels of the previous one, and accumulates every
+ * chunk into the same O(K D) statistics (the chunked scheme the paper's Limitations section describes).
+ * All other arrays are host pointers too.  Synchronises the stream. */
+int gmm_em_step_host(gmm_ctx* ctx, const float* X_host, int64_t N, int D, int K,
+                     const float* pi_host, const float* mu_host, const float* var_host,
+                     double* Nk_host, double* S1_host, double* S2_host, double* loglik);
+
+/* Parameter update from the statistics (paper Section 2: pi_k = N_k / N; Eq. 2; Eq. 3 taken per dimension with the
+ * new mean, i.e. var_kd = max(S2_kd / N_k - mu_kd^2, var_floor); Algorithm 1's last line).
+ *   Nk, S1, S2 device float64 inputs; pi, mu, var device float32, in/out: a component with N_k < 1e-12 keeps its
+ *   mu and var (its pi becomes N_k / N).  Asynchronous on the stream. */
+int gmm_finalize(gmm_ctx* ctx, int64_t N, int D, int K,
+                 const double* Nk, const double* S1, const double* S2,
+                 float var_floor, float* pi, float* mu, float* var);
+
+/* EM driver: `iters` iterations of gmm_em_step + gmm_finalize (paper Section 2, last paragraph; Algorithm 1 run
+ * repeatedly).  pi/mu/var: device, in = initial parameters, out = fitted.  loglik_trace: host [iters];
+ * trace[t] is the log-likelihood under the parameters ENTERING iteration t.  tol > 0 stops after iteration t >= 1
+ * when |L_t - L_{t-1}| <= tol * |L_t|; tol = 0 runs all iterations.  iters_done (host, may be NULL) receives the
+ * number of iterations run.  Synchronises the stream. */
+int gmm_fit(gmm_ctx* ctx, const float* X, int64_t N, int D, int K,
+            float* pi, float* mu, float* var,
+            int iters, float var_floor, double tol,
+            double* loglik_trace, int* iters_done);
+
+/* Top-m components by responsibility for every point (paper Section 4.2: the arg-max assignment; Section 4.3: the
+ * clusters with the largest responsibilities, which the caller thresholds with tau = 1/K).
+ *   idx [N x m] int32 and resp [N x m] float32, device outputs; per point descending by responsibility, ties to the
+ *   smaller component index.  1 <= m <= min(K, GMM_MAX_TOPM).  Asynchronous on the stream. */
+int gmm_assign_topm(gmm_ctx* ctx, const float* X, int64_t N, int D, int K,
+                    const float* pi, const float* mu, const float* var, int m,
+                    int32_t* idx, float* resp);
+
+/* Bytes of device scratch a context holds for shape (D, K); independent of N. */
+size_t gmm_scratch_bytes(int D, int K);
+
+/* Instrumentation.  Kernel launches enqueued by this context since creation (or the last reset). */
+int64_t gmm_launch_count(const gmm_ctx* ctx);
+/* With profiling on, the dominant kernel of each compute call (the E/M tile kernel) is bracketed by CUDA events on
+ * the context's stream.  gmm_kernel_time synchronises the stream and returns the summed event time in
+ * milliseconds and the number of bracketed launches since the last gmm_reset_counters. */
+int gmm_set_profiling(gmm_ctx* ctx, int on);
+int gmm_kernel_time(gmm_ctx* ctx, double* total_ms, int64_t* launches);
+int gmm_reset_counters(gmm_ctx* ctx);
+
+const char* gmm_strerror(int code);
+const char* gmm_last_error(const gmm_ctx* ctx);
+const char* gmm_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FLASHGMM_H */

@@ -1,0 +1,420 @@
+// FP32 CUDA-core path: direct differences (x - mu)^2 / var, two phases per super-tile of points.
+//
+// Phase 1 (lse_kernel): for a tile of 64 points sweep all K components in blocks of 64, keep the running
+//   (max, sum) of the online log-sum-exp per point on chip, write log Z_i (paper Algorithm 1, Step 1).
+// Phase 2 (mstep_kernel): a CTA owns 64 components (and a 128-wide slice of D); for each of its point tiles it
+//   recomputes log z_ik, forms r_ik = exp(log z_ik - log Z_i) in shared memory and accumulates N_k, S1, S2 in
+//   registers across ALL its tiles (Algorithm 1, Step 2) -- the accumulators leave the SM once, as a per-CTA
+//   partial; there are no atomics.
+// The arithmetic is in the log2 domain: w2 = (log2 e / 2) / var, c2 = log2 e * (log pi - 1/2 sum_d log(2 pi var)),
+// log2 z = c2 - sum_d w2 (x - mu)^2, so the exponential is a bare ex2.
+#include "internal.cuh"
+#include <math_constants.h>
+
+namespace fg {
+
+namespace {
+
+constexpr int TP = FP32_TILE_P;
+constexpr int TC = FP32_TILE_C;
+constexpr int DCH = 32;       // dimensions staged per step
+constexpr int LDT = 68;       // shared-memory row stride in floats (16-byte aligned rows, fewer store conflicts)
+constexpr int NTHREADS = 256;
+
+struct TileSmem {
+    float xs[DCH][LDT];
+    float ms[DCH][LDT];
+    float ws[DCH][LDT];
+};
+
+__device__ __forceinline__ float fast_ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// q[a][b] = sum_d w2[k0 + 4 tx + b][d] * (X[row0 + 4 ty + a][d] - mu[k0 + 4 tx + b][d])^2
+// Rows >= n and components >= K are staged as zeros (w2 = 0 -> contributes nothing).
+__device__ __forceinline__ void tile_quadratic(TileSmem& sm, const float* __restrict__ X, int64_t row0, int64_t n,
+                                               int D, const float* __restrict__ mu, const float* __restrict__ w2,
+                                               int k0, int K, float (&q)[4][4]) {
+    const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) q[a][b] = 0.f;
+    for (int d0 = 0; d0 < D; d0 += DCH) {
+        __syncthreads();
+#pragma unroll
+        for (int j = 0; j < (TP * DCH) / NTHREADS; ++j) {
+            const int e = tid + j * NTHREADS, r = e >> 5, c = e & 31, d = d0 + c;
+            const int64_t row = row0 + r;
+            const int k = k0 + r;
+            float xv = 0.f, mv = 0.f, wv = 0.f;
+            if (d < D) {
+                if (row < n) xv = __ldg(X + row * D + d);
+                if (k < K) {
+                    mv = __ldg(mu + (size_t)k * D + d);
+                    wv = __ldg(w2 + (size_t)k * D + d);
+                }
+            }
+            sm.xs[c][r] = xv;
+            sm.ms[c][r] = mv;
+            sm.ws[c][r] = wv;
+        }
+        __syncthreads();
+#pragma unroll 8
+        for (int c = 0; c < DCH; ++c) {
+            const float4 xv = *reinterpret_cast<const float4*>(&sm.xs[c][4 * ty]);
+            const float4 mv = *reinterpret_cast<const float4*>(&sm.ms[c][4 * tx]);
+            const float4 wv = *reinterpret_cast<const float4*>(&sm.ws[c][4 * tx]);
+            const float xa[4] = {xv.x, xv.y, xv.z, xv.w};
+            const float mb[4] = {mv.x, mv.y, mv.z, mv.w};
+            const float wb[4] = {wv.x, wv.y, wv.z, wv.w};
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+#pragma unroll
+                for (int b = 0; b < 4; ++b) {
+                    const float diff = xa[a] - mb[b];
+                    q[a][b] = fmaf(diff * diff, wb[b], q[a][b]);
+                }
+        }
+    }
+}
+
+template <int M>
+struct TopList {
+    float v[M];
+    int i[M];
+    __device__ __forceinline__ void init() {
+#pragma unroll
+        for (int j = 0; j < M; ++j) { v[j] = -CUDART_INF_F; i[j] = -1; }
+    }
+    // insert keeping descending order; equal values keep the earlier (smaller) index first
+    __device__ __forceinline__ void insert(float val, int id) {
+        if (i[M - 1] >= 0 && !(val > v[M - 1])) return;
+        v[M - 1] = val; i[M - 1] = id;
+#pragma unroll
+        for (int j = M - 1; j > 0; --j) {
+            const bool up = (i[j - 1] < 0) || (v[j] > v[j - 1]);
+            if (up) {
+                const float tv = v[j]; v[j] = v[j - 1]; v[j - 1] = tv;
+                const int ti = i[j]; i[j] = i[j - 1]; i[j - 1] = ti;
+            }
+        }
+    }
+};
+
+// M == 0: log-sum-exp only.  M > 0: also the top-M components per point.
+template <int M>
+__global__ void __launch_bounds__(NTHREADS)
+lse_kernel(const float* __restrict__ X, int64_t n, int D, int K, const float* __restrict__ mu,
+           const float* __restrict__ w2, const float* __restrict__ c2, float* __restrict__ logZ2,
+           double* __restrict__ llpart, int m_out, int32_t* __restrict__ idx_out, float* __restrict__ resp_out) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    TileSmem& sm = *reinterpret_cast<TileSmem*>(smem_raw);
+    __shared__ double ll_s[TP];
+    const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+    const int64_t row0 = (int64_t)blockIdx.x * TP;
+
+    float m_run[4], s_run[4];
+#pragma unroll
+    for (int a = 0; a < 4; ++a) { m_run[a] = -CUDART_INF_F; s_run[a] = 0.f; }
+    TopList<(M > 0 ? M : 1)> top[4];
+    if (M > 0) {
+#pragma unroll
+        for (int a = 0; a < 4; ++a) top[a].init();
+    }
+
+    for (int k0 = 0; k0 < K; k0 += TC) {
+        float q[4][4];
+        tile_quadratic(sm, X, row0, n, D, mu, w2, k0, K, q);
+        float cv[4];
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            const int k = k0 + 4 * tx + b;
+            cv[b] = (k < K) ? __ldg(c2 + k) : -CUDART_INF_F;
+        }
+#pragma unroll
+        for (int a = 0; a < 4; ++a) {
+            float l[4];
+#pragma unroll
+            for (int b = 0; b < 4; ++b) l[b] = cv[b] - q[a][b];
+            if (M > 0) {
+#pragma unroll
+                for (int b = 0; b < 4; ++b)
+                    if (k0 + 4 * tx + b < K) top[a].insert(l[b], k0 + 4 * tx + b);
+            }
+            float mloc = fmaxf(fmaxf(l[0], l[1]), fmaxf(l[2], l[3]));
+#pragma unroll
+            for (int o = 8; o > 0; o >>= 1) mloc = fmaxf(mloc, __shfl_xor_sync(0xffffffffu, mloc, o));
+            const float m_new = fmaxf(m_run[a], mloc);
+            const float m_safe = (m_new == -CUDART_INF_F) ? 0.f : m_new;
+            float sloc = fast_ex2(l[0] - m_safe) + fast_ex2(l[1] - m_safe) + fast_ex2(l[2] - m_safe) +
+                         fast_ex2(l[3] - m_safe);
+#pragma unroll
+            for (int o = 8; o > 0; o >>= 1) sloc += __shfl_xor_sync(0xffffffffu, sloc, o);
+            s_run[a] = s_run[a] * fast_ex2(m_run[a] - m_safe) + sloc;
+            m_run[a] = m_new;
+        }
+    }
+
+    float lz[4];
+#pragma unroll
+    for (int a = 0; a < 4; ++a) lz[a] = m_run[a] + log2f(s_run[a]);
+    if (tx == 0) {
+#pragma unroll
+        for (int a = 0; a < 4; ++a) {
+            const int64_t row = row0 + 4 * ty + a;
+            const bool ok = row < n;
+            if (ok && logZ2) logZ2[row] = lz[a];
+            ll_s[4 * ty + a] = ok ? (double)lz[a] * 0.69314718055994530942 : 0.0;
+        }
+    }
+    if (M > 0) {
+        // merge the 16 per-thread lists of each point through shared memory (reuses the staging area)
+        __syncthreads();
+        float* cand_v = reinterpret_cast<float*>(smem_raw);
+        int* cand_i = reinterpret_cast<int*>(smem_raw) + TP * 16 * M;
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+#pragma unroll
+            for (int j = 0; j < M; ++j) {
+                const int slot = (4 * ty + a) * 16 * M + tx * M + j;
+                cand_v[slot] = top[a].v[j];
+                cand_i[slot] = top[a].i[j];
+            }
+        __shared__ float lz_s[TP];
+        if (tx == 0) {
+#pragma unroll
+            for (int a = 0; a < 4; ++a) lz_s[4 * ty + a] = lz[a];
+        }
+        __syncthreads();
+        if (tid < TP && row0 + tid < n) {
+            float* cv = cand_v + tid * 16 * M;
+            int* ci = cand_i + tid * 16 * M;
+            const float lzp = lz_s[tid];
+            for (int j = 0; j < m_out; ++j) {
+                int best = -1;
+                for (int s = 0; s < 16 * M; ++s) {
+                    if (ci[s] < 0) continue;
+                    if (best < 0 || cv[s] > cv[best] || (cv[s] == cv[best] && ci[s] < ci[best])) best = s;
+                }
+                int id = 0;
+                float r = 0.f;
+                if (best >= 0) {
+                    id = ci[best];
+                    r = fast_ex2(cv[best] - lzp);
+                    ci[best] = -1;
+                }
+                idx_out[(row0 + tid) * m_out + j] = id;
+                resp_out[(row0 + tid) * m_out + j] = r;
+            }
+        }
+    }
+    if (llpart) {
+        __syncthreads();
+        if (tid == 0) {
+            double s = 0.0;
+            for (int i = 0; i < TP; ++i) s += ll_s[i];
+            llpart[blockIdx.x] = s;
+        }
+    }
+}
+
+constexpr int LDR = TC + 4;                 // r tile row stride
+constexpr int LDX = FP32_MSTEP_DC + 4;      // X tile row stride
+constexpr size_t MSTEP_SMEM = sizeof(TileSmem) + (size_t)TP * LDR * 4 + (size_t)TP * LDX * 4;
+
+__global__ void __launch_bounds__(NTHREADS)
+mstep_kernel(const float* __restrict__ X, int64_t n, int D, int K, const float* __restrict__ mu,
+             const float* __restrict__ w2, const float* __restrict__ c2, const float* __restrict__ logZ2,
+             float* __restrict__ partials) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    TileSmem& sm = *reinterpret_cast<TileSmem*>(smem_raw);
+    float* r_s = reinterpret_cast<float*>(smem_raw + sizeof(TileSmem));     // [TP][LDR]
+    float* xm = r_s + TP * LDR;                                              // [TP][LDX]
+    const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+    const int kq = tid >> 5, dq = tid & 31;
+    const int k0 = blockIdx.x * TC;
+    const int split = blockIdx.y, nsplits = gridDim.y;
+    const int dz0 = blockIdx.z * FP32_MSTEP_DC;
+    const int64_t ntiles = (n + TP - 1) / TP;
+
+    float acc1[8][4], acc2[8][4];
+#pragma unroll
+    for (int c = 0; c < 8; ++c)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { acc1[c][j] = 0.f; acc2[c][j] = 0.f; }
+    float nacc = 0.f;
+    float cv[4];
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+        const int k = k0 + 4 * tx + b;
+        cv[b] = (k < K) ? __ldg(c2 + k) : -CUDART_INF_F;
+    }
+
+    for (int64_t t = split; t < ntiles; t += nsplits) {
+        const int64_t row0 = t * TP;
+        float q[4][4];
+        tile_quadratic(sm, X, row0, n, D, mu, w2, k0, K, q);
+#pragma unroll
+        for (int a = 0; a < 4; ++a) {
+            const int64_t row = row0 + 4 * ty + a;
+            const float lz = (row < n) ? __ldg(logZ2 + row) : CUDART_INF_F;    // +inf -> r = 0 for padded rows
+            float4 rv;
+            rv.x = fast_ex2(cv[0] - q[a][0] - lz);
+            rv.y = fast_ex2(cv[1] - q[a][1] - lz);
+            rv.z = fast_ex2(cv[2] - q[a][2] - lz);
+            rv.w = fast_ex2(cv[3] - q[a][3] - lz);
+            *reinterpret_cast<float4*>(&r_s[(4 * ty + a) * LDR + 4 * tx]) = rv;
+        }
+        // stage this CTA's D-slice of the X tile, row-major
+#pragma unroll 4
+        for (int j = 0; j < (TP * FP32_MSTEP_DC) / NTHREADS; ++j) {
+            const int e = tid + j * NTHREADS, r = e >> 7, c = e & 127;
+            const int64_t row = row0 + r;
+            const int d = dz0 + c;
+            xm[r * LDX + c] = (row < n && d < D) ? __ldg(X + row * D + d) : 0.f;
+        }
+        __syncthreads();
+        if (tid < TC) {
+            float s = 0.f;
+#pragma unroll 8
+            for (int i = 0; i < TP; ++i) s += r_s[i * LDR + tid];
+            nacc += s;
+        }
+#pragma unroll 2
+        for (int i = 0; i < TP; ++i) {
+            const float4 xv = *reinterpret_cast<const float4*>(&xm[i * LDX + 4 * dq]);
+            const float4 ra = *reinterpret_cast<const float4*>(&r_s[i * LDR + 8 * kq]);
+            const float4 rb = *reinterpret_cast<const float4*>(&r_s[i * LDR + 8 * kq + 4]);
+            const float x1[4] = {xv.x, xv.y, xv.z, xv.w};
+            const float x2[4] = {xv.x * xv.x, xv.y * xv.y, xv.z * xv.z, xv.w * xv.w};
+            const float rr[8] = {ra.x, ra.y, ra.z, ra.w, rb.x, rb.y, rb.z, rb.w};
+#pragma unroll
+            for (int c = 0; c < 8; ++c)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    acc1[c][j] = fmaf(rr[c], x1[j], acc1[c][j]);
+                    acc2[c][j] = fmaf(rr[c], x2[j], acc2[c][j]);
+                }
+        }
+        // the next tile_quadratic starts with __syncthreads(), which also protects r_s / xm
+    }
+
+    const size_t KD = (size_t)K * D;
+    float* pN = partials + (size_t)split * (K + 2 * KD);
+    float* pS1 = pN + K;
+    float* pS2 = pS1 + KD;
+    if (blockIdx.z == 0 && tid < TC && k0 + tid < K) pN[k0 + tid] = nacc;
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+        const int k = k0 + 8 * kq + c;
+        if (k >= K) continue;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int d = dz0 + 4 * dq + j;
+            if (d < D) {
+                pS1[(size_t)k * D + d] = acc1[c][j];
+                pS2[(size_t)k * D + d] = acc2[c][j];
+            }
+        }
+    }
+}
+
+// One block per component: w2 = (log2 e / 2) / var, c2 = log2 e (log pi - 1/2 sum_d log(2 pi var)), in float64.
+__global__ void prepare_fp32_kernel(int D, int K, const float* __restrict__ pi, const float* __restrict__ mu,
+                                    const float* __restrict__ var, float* __restrict__ w2, float* __restrict__ c2,
+                                    int* __restrict__ status) {
+    const int k = blockIdx.x;
+    __shared__ double red[128];
+    double s = 0.0;
+    int bad = 0;
+    for (int d = threadIdx.x; d < D; d += blockDim.x) {
+        const float v = var[(size_t)k * D + d];
+        const float m = mu[(size_t)k * D + d];
+        if (!(v > 0.f) || !isfinite(v)) bad |= ST_BAD_VAR;
+        if (!isfinite(m)) bad |= ST_NONFINITE;
+        const double vd = (double)v;
+        s += log(6.283185307179586476925286766559 * vd);
+        w2[(size_t)k * D + d] = (float)(0.72134752044448170368 / vd);
+    }
+    red[threadIdx.x] = s;
+    __syncthreads();
+    for (int o = blockDim.x / 2; o > 0; o >>= 1) {
+        if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        const float p = pi[k];
+        if (!(p >= 0.f) || !isfinite(p)) bad |= ST_BAD_PI;
+        const double lp = (p > 0.f) ? log((double)p) : -CUDART_INF;
+        c2[k] = (float)(1.4426950408889634074 * (lp - 0.5 * red[0]));
+    }
+    if (bad) atomicOr(status, bad);
+}
+
+}  // namespace
+
+Fp32Plan fp32_plan(int D, int K) {
+    Fp32Plan p;
+    p.comp_blocks = (K + TC - 1) / TC;
+    p.d_chunks = (D + FP32_MSTEP_DC - 1) / FP32_MSTEP_DC;
+    const int per = p.comp_blocks * p.d_chunks;
+    p.splits = (FP32_TARGET_CTAS + per - 1) / per;
+    if (p.splits < 1) p.splits = 1;
+    return p;
+}
+
+size_t fp32_partial_floats(int D, int K) {
+    const Fp32Plan p = fp32_plan(D, K);
+    return (size_t)p.splits * ((size_t)K + 2 * (size_t)K * D);
+}
+
+cudaError_t launch_prepare_fp32(cudaStream_t s, int D, int K, const float* pi, const float* mu, const float* var,
+                                float* w2, float* c2, int* status) {
+    prepare_fp32_kernel<<<K, 128, 0, s>>>(D, K, pi, mu, var, w2, c2, status);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_lse_fp32(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu,
+                            const float* w2, const float* c2, float* logZ2, double* llpart) {
+    const unsigned blocks = (unsigned)((n + TP - 1) / TP);
+    lse_kernel<0><<<blocks, NTHREADS, sizeof(TileSmem), s>>>(X, n, D, K, mu, w2, c2, logZ2, llpart, 0, nullptr,
+                                                            nullptr);
+    return cudaGetLastError();
+}
+
+template <int M>
+static cudaError_t launch_topm_t(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu,
+                                 const float* w2, const float* c2, int m, int32_t* idx, float* resp) {
+    size_t smem = sizeof(TileSmem);
+    const size_t need = (size_t)TP * 16 * M * 8;
+    if (need > smem) smem = need;
+    cudaError_t e = cudaFuncSetAttribute(lse_kernel<M>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    const unsigned blocks = (unsigned)((n + TP - 1) / TP);
+    lse_kernel<M><<<blocks, NTHREADS, smem, s>>>(X, n, D, K, mu, w2, c2, nullptr, nullptr, m, idx, resp);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_topm_fp32(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu,
+                             const float* w2, const float* c2, int m, int32_t* idx, float* resp) {
+    if (m <= 1) return launch_topm_t<1>(s, X, n, D, K, mu, w2, c2, m, idx, resp);
+    if (m <= 2) return launch_topm_t<2>(s, X, n, D, K, mu, w2, c2, m, idx, resp);
+    if (m <= 4) return launch_topm_t<4>(s, X, n, D, K, mu, w2, c2, m, idx, resp);
+    return launch_topm_t<8>(s, X, n, D, K, mu, w2, c2, m, idx, resp);
+}
+
+cudaError_t launch_mstep_fp32(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu,
+                              const float* w2, const float* c2, const float* logZ2, float* partials,
+                              const Fp32Plan& plan) {
+    cudaError_t e = cudaFuncSetAttribute(mstep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)MSTEP_SMEM);
+    if (e != cudaSuccess) return e;
+    dim3 grid(plan.comp_blocks, plan.splits, plan.d_chunks);
+    mstep_kernel<<<grid, NTHREADS, MSTEP_SMEM, s>>>(X, n, D, K, mu, w2, c2, logZ2, partials);
+    return cudaGetLastError();
+}
+
+}  // namespace fg

@@ -1,0 +1,538 @@
+// Host side of libflashgmm: context, argument checking, scratch management, path dispatch, the EM driver and the
+// host-streaming variant.  Every step of the numerical path runs in the CUDA kernels of the other files.
+#include "internal.cuh"
+
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+using namespace fg;
+
+namespace {
+
+struct DevResult {
+    double ll[LL_SLOTS];
+    int status;
+    int pad;
+};
+
+constexpr size_t STAGE_BYTES = (size_t)128 << 20;   // per staging buffer of the host-streaming path
+constexpr int EVENT_POOL = 128;
+
+inline size_t align256(size_t b) { return (b + 255) & ~(size_t)255; }
+
+struct ScratchLayout {
+    size_t w2, c2, partials, logZ2, llpart, result, stats, derived_tc, total;
+};
+
+ScratchLayout scratch_layout(int D, int K) {
+    ScratchLayout L;
+    const size_t KD = (size_t)K * D;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off += align256(bytes); return o; };
+    L.w2 = take(KD * 4);
+    L.c2 = take((size_t)K * 4);
+    L.partials = take(fp32_partial_floats(D, K) * 4);
+    L.logZ2 = take((size_t)SUPER_TILE * 4);
+    L.llpart = take((size_t)(SUPER_TILE / FP32_TILE_P) * 8);
+    L.result = take(sizeof(DevResult));
+    L.stats = take(((size_t)K + 2 * KD) * 8);
+    L.derived_tc = take(0);
+    L.total = off;
+    return L;
+}
+
+}  // namespace
+
+struct gmm_ctx {
+    int device = 0;
+    cudaStream_t stream = nullptr;
+    int path = GMM_PATH_AUTO;
+    int last_path = 0;
+    // scratch
+    unsigned char* scratch = nullptr;
+    size_t scratch_bytes = 0;
+    int capD = 0, capK = 0;
+    ScratchLayout lay{};
+    // host-streaming path
+    cudaStream_t copy_stream = nullptr;
+    float* xstage[2] = {nullptr, nullptr};
+    cudaEvent_t ev_copied[2] = {nullptr, nullptr}, ev_done[2] = {nullptr, nullptr};
+    float* hparams = nullptr;      // device copies of pi, mu, var for the host path
+    size_t hparams_floats = 0;
+    // instrumentation
+    int64_t launches = 0;
+    bool profiling = false;
+    cudaEvent_t ev_a[EVENT_POOL], ev_b[EVENT_POOL];
+    int ev_used = 0;
+    bool ev_created = false;
+    double prof_ms = 0.0;
+    int64_t prof_launches = 0;
+    char err[512] = {0};
+
+    float* w2() const { return reinterpret_cast<float*>(scratch + lay.w2); }
+    float* c2() const { return reinterpret_cast<float*>(scratch + lay.c2); }
+    float* partials() const { return reinterpret_cast<float*>(scratch + lay.partials); }
+    float* logZ2() const { return reinterpret_cast<float*>(scratch + lay.logZ2); }
+    double* llpart() const { return reinterpret_cast<double*>(scratch + lay.llpart); }
+    DevResult* result() const { return reinterpret_cast<DevResult*>(scratch + lay.result); }
+    double* stats() const { return reinterpret_cast<double*>(scratch + lay.stats); }
+};
+
+namespace {
+
+int fail(gmm_ctx* ctx, int code, const char* fmt, ...) {
+    if (ctx) {
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(ctx->err, sizeof(ctx->err), fmt, ap);
+        va_end(ap);
+    }
+    return code;
+}
+
+#define CU(call)                                                                                      \
+    do {                                                                                              \
+        cudaError_t e_ = (call);                                                                      \
+        if (e_ != cudaSuccess)                                                                        \
+            return fail(ctx, GMM_ECUDA, "%s failed: %s (%s:%d)", #call, cudaGetErrorString(e_), __FILE__, __LINE__); \
+    } while (0)
+
+#define KL(call)                                                                                      \
+    do {                                                                                              \
+        cudaError_t e_ = (call);                                                                      \
+        if (e_ != cudaSuccess)                                                                        \
+            return fail(ctx, GMM_ECUDA, "%s failed: %s (%s:%d)", #call, cudaGetErrorString(e_), __FILE__, __LINE__); \
+        ctx->launches++;                                                                              \
+    } while (0)
+
+int ensure_scratch(gmm_ctx* ctx, int D, int K) {
+    if (ctx->scratch && D == ctx->capD && K == ctx->capK) return GMM_OK;
+    const ScratchLayout L = scratch_layout(D, K);
+    if (L.total > ctx->scratch_bytes) {
+        if (ctx->scratch) {
+            CU(cudaStreamSynchronize(ctx->stream));
+            CU(cudaFree(ctx->scratch));
+            ctx->scratch = nullptr;
+            ctx->scratch_bytes = 0;
+        }
+        void* p = nullptr;
+        cudaError_t e = cudaMalloc(&p, L.total);
+        if (e != cudaSuccess) {
+            cudaGetLastError();
+            return fail(ctx, GMM_ENOMEM, "cannot allocate %zu bytes of scratch: %s", L.total, cudaGetErrorString(e));
+        }
+        ctx->scratch = static_cast<unsigned char*>(p);
+        ctx->scratch_bytes = L.total;
+    }
+    ctx->lay = L;
+    ctx->capD = D;
+    ctx->capK = K;
+    return GMM_OK;
+}
+
+int check_shape(gmm_ctx* ctx, int64_t N, int D, int K) {
+    if (!ctx) return GMM_EINVAL;
+    if (N < 1 || D < 1 || K < 1) return fail(ctx, GMM_EINVAL, "N, D and K must be >= 1 (got N=%lld D=%d K=%d)", (long long)N, D, K);
+    if ((int64_t)K * D > ((int64_t)1 << 28)) return fail(ctx, GMM_EINVAL, "K*D too large (%lld)", (long long)K * D);
+    return GMM_OK;
+}
+
+int check_ptr(gmm_ctx* ctx, const void* p, size_t align, const char* name) {
+    if (!p) return fail(ctx, GMM_EINVAL, "%s is NULL", name);
+    if (reinterpret_cast<uintptr_t>(p) % align) return fail(ctx, GMM_EALIGN, "%s is not %zu-byte aligned", name, align);
+    return GMM_OK;
+}
+
+#define CHECK(expr)            \
+    do {                       \
+        int rc_ = (expr);      \
+        if (rc_ != GMM_OK) return rc_; \
+    } while (0)
+
+int prof_begin(gmm_ctx* ctx) {
+    if (!ctx->profiling) return GMM_OK;
+    if (!ctx->ev_created) {
+        for (int i = 0; i < EVENT_POOL; ++i) {
+            CU(cudaEventCreate(&ctx->ev_a[i]));
+            CU(cudaEventCreate(&ctx->ev_b[i]));
+        }
+        ctx->ev_created = true;
+    }
+    if (ctx->ev_used == EVENT_POOL) {
+        CU(cudaStreamSynchronize(ctx->stream));
+        for (int i = 0; i < ctx->ev_used; ++i) {
+            float ms = 0.f;
+            CU(cudaEventElapsedTime(&ms, ctx->ev_a[i], ctx->ev_b[i]));
+            ctx->prof_ms += ms;
+        }
+        ctx->ev_used = 0;
+    }
+    CU(cudaEventRecord(ctx->ev_a[ctx->ev_used], ctx->stream));
+    return GMM_OK;
+}
+
+int prof_end(gmm_ctx* ctx) {
+    if (!ctx->profiling) return GMM_OK;
+    CU(cudaEventRecord(ctx->ev_b[ctx->ev_used], ctx->stream));
+    ctx->ev_used++;
+    ctx->prof_launches++;
+    return GMM_OK;
+}
+
+int choose_path(gmm_ctx* ctx, int D, int K, int* path) {
+    (void)D; (void)K;
+    if (ctx->path == GMM_PATH_TENSOR) return fail(ctx, GMM_EUNSUPPORTED, "the tensor-core path cannot run D=%d K=%d", D, K);
+    *path = GMM_PATH_FP32;
+    return GMM_OK;
+}
+
+// Derived per-component constants for the chosen path; validates the parameters into the status word.
+int prepare_params(gmm_ctx* ctx, int path, int D, int K, const float* pi, const float* mu, const float* var) {
+    (void)path;
+    CU(cudaMemsetAsync(&ctx->result()->status, 0, sizeof(int), ctx->stream));
+    KL(launch_prepare_fp32(ctx->stream, D, K, pi, mu, var, ctx->w2(), ctx->c2(), &ctx->result()->status));
+    return GMM_OK;
+}
+
+// Adds the statistics of n device-resident points to (Nk, S1, S2) and their log-likelihood to result()->ll[slot].
+int accumulate_points(gmm_ctx* ctx, int path, const float* X, int64_t n, int D, int K, const float* mu, double* Nk,
+                      double* S1, double* S2, int slot) {
+    (void)path;
+    const Fp32Plan plan = fp32_plan(D, K);
+    for (int64_t off = 0; off < n; off += SUPER_TILE) {
+        const int64_t cnt = (n - off < SUPER_TILE) ? (n - off) : SUPER_TILE;
+        const float* Xs = X + off * D;
+        CHECK(prof_begin(ctx));
+        KL(launch_lse_fp32(ctx->stream, Xs, cnt, D, K, mu, ctx->w2(), ctx->c2(), ctx->logZ2(), ctx->llpart()));
+        KL(launch_mstep_fp32(ctx->stream, Xs, cnt, D, K, mu, ctx->w2(), ctx->c2(), ctx->logZ2(), ctx->partials(), plan));
+        CHECK(prof_end(ctx));
+        KL(launch_reduce_ll(ctx->stream, ctx->llpart(), (cnt + FP32_TILE_P - 1) / FP32_TILE_P, &ctx->result()->ll[slot], true));
+        KL(launch_reduce_partials(ctx->stream, D, K, plan.splits, ctx->partials(), Nk, S1, S2, true));
+    }
+    return GMM_OK;
+}
+
+int zero_stats(gmm_ctx* ctx, int D, int K, double* Nk, double* S1, double* S2, int slot) {
+    const size_t KD = (size_t)K * D;
+    CU(cudaMemsetAsync(Nk, 0, (size_t)K * 8, ctx->stream));
+    CU(cudaMemsetAsync(S1, 0, KD * 8, ctx->stream));
+    CU(cudaMemsetAsync(S2, 0, KD * 8, ctx->stream));
+    CU(cudaMemsetAsync(&ctx->result()->ll[slot], 0, 8, ctx->stream));
+    return GMM_OK;
+}
+
+// Synchronising read of the log-likelihood slot and the status word.
+int read_result(gmm_ctx* ctx, int slot, double* loglik) {
+    DevResult r;
+    CU(cudaMemcpyAsync(&r, ctx->result(), sizeof(DevResult), cudaMemcpyDeviceToHost, ctx->stream));
+    CU(cudaStreamSynchronize(ctx->stream));
+    if (r.status & ST_TIMEOUT) return fail(ctx, GMM_ETIMEOUT, "a bounded device-side wait expired");
+    if (r.status & ST_BAD_VAR) return fail(ctx, GMM_ENUMERIC, "var must be finite and > 0");
+    if (r.status & ST_BAD_PI) return fail(ctx, GMM_ENUMERIC, "pi must be finite and >= 0");
+    if (r.status & ST_NONFINITE) return fail(ctx, GMM_ENUMERIC, "non-finite parameter");
+    *loglik = r.ll[slot];
+    if (!std::isfinite(*loglik)) return fail(ctx, GMM_ENUMERIC, "log-likelihood is not finite (%g)", *loglik);
+    return GMM_OK;
+}
+
+struct DeviceGuard {
+    int prev = -1;
+    explicit DeviceGuard(int dev) {
+        cudaGetDevice(&prev);
+        if (prev != dev) cudaSetDevice(dev);
+        else prev = -1;
+    }
+    ~DeviceGuard() {
+        if (prev >= 0) cudaSetDevice(prev);
+    }
+};
+
+}  // namespace
+
+extern "C" {
+
+int gmm_create(gmm_ctx** out, int device, void* cuda_stream) {
+    if (!out) return GMM_EINVAL;
+    *out = nullptr;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) {
+        cudaGetLastError();
+        return GMM_ECUDA;
+    }
+    gmm_ctx* ctx = new (std::nothrow) gmm_ctx();
+    if (!ctx) return GMM_ENOMEM;
+    ctx->device = device;
+    ctx->stream = static_cast<cudaStream_t>(cuda_stream);
+    *out = ctx;
+    return GMM_OK;
+}
+
+int gmm_destroy(gmm_ctx* ctx) {
+    if (!ctx) return GMM_EINVAL;
+    DeviceGuard g(ctx->device);
+    cudaStreamSynchronize(ctx->stream);
+    if (ctx->scratch) cudaFree(ctx->scratch);
+    for (int b = 0; b < 2; ++b) {
+        if (ctx->xstage[b]) cudaFree(ctx->xstage[b]);
+        if (ctx->ev_copied[b]) cudaEventDestroy(ctx->ev_copied[b]);
+        if (ctx->ev_done[b]) cudaEventDestroy(ctx->ev_done[b]);
+    }
+    if (ctx->hparams) cudaFree(ctx->hparams);
+    if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
+    if (ctx->ev_created)
+        for (int i = 0; i < EVENT_POOL; ++i) {
+            cudaEventDestroy(ctx->ev_a[i]);
+            cudaEventDestroy(ctx->ev_b[i]);
+        }
+    cudaGetLastError();
+    delete ctx;
+    return GMM_OK;
+}
+
+int gmm_set_path(gmm_ctx* ctx, int path) {
+    if (!ctx) return GMM_EINVAL;
+    if (path != GMM_PATH_AUTO && path != GMM_PATH_FP32 && path != GMM_PATH_TENSOR)
+        return fail(ctx, GMM_EINVAL, "unknown path %d", path);
+    ctx->path = path;
+    return GMM_OK;
+}
+
+int gmm_last_path(const gmm_ctx* ctx) { return ctx ? ctx->last_path : GMM_EINVAL; }
+
+int gmm_em_step(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const float* pi, const float* mu,
+                const float* var, double* Nk, double* S1, double* S2, double* loglik) {
+    CHECK(check_shape(ctx, N, D, K));
+    CHECK(check_ptr(ctx, X, 4, "X"));
+    CHECK(check_ptr(ctx, pi, 4, "pi"));
+    CHECK(check_ptr(ctx, mu, 4, "mu"));
+    CHECK(check_ptr(ctx, var, 4, "var"));
+    CHECK(check_ptr(ctx, Nk, 8, "Nk"));
+    CHECK(check_ptr(ctx, S1, 8, "S1"));
+    CHECK(check_ptr(ctx, S2, 8, "S2"));
+    if (!loglik) return fail(ctx, GMM_EINVAL, "loglik is NULL");
+    DeviceGuard g(ctx->device);
+    int path;
+    CHECK(choose_path(ctx, D, K, &path));
+    CHECK(ensure_scratch(ctx, D, K));
+    CHECK(prepare_params(ctx, path, D, K, pi, mu, var));
+    CHECK(zero_stats(ctx, D, K, Nk, S1, S2, 0));
+    CHECK(accumulate_points(ctx, path, X, N, D, K, mu, Nk, S1, S2, 0));
+    ctx->last_path = path;
+    return read_result(ctx, 0, loglik);
+}
+
+int gmm_finalize(gmm_ctx* ctx, int64_t N, int D, int K, const double* Nk, const double* S1, const double* S2,
+                 float var_floor, float* pi, float* mu, float* var) {
+    CHECK(check_shape(ctx, N, D, K));
+    CHECK(check_ptr(ctx, Nk, 8, "Nk"));
+    CHECK(check_ptr(ctx, S1, 8, "S1"));
+    CHECK(check_ptr(ctx, S2, 8, "S2"));
+    CHECK(check_ptr(ctx, pi, 4, "pi"));
+    CHECK(check_ptr(ctx, mu, 4, "mu"));
+    CHECK(check_ptr(ctx, var, 4, "var"));
+    if (!(var_floor >= 0.f)) return fail(ctx, GMM_EINVAL, "var_floor must be >= 0");
+    DeviceGuard g(ctx->device);
+    KL(launch_finalize(ctx->stream, N, D, K, Nk, S1, S2, var_floor, pi, mu, var));
+    return GMM_OK;
+}
+
+int gmm_fit(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, float* pi, float* mu, float* var, int iters,
+            float var_floor, double tol, double* loglik_trace, int* iters_done) {
+    CHECK(check_shape(ctx, N, D, K));
+    CHECK(check_ptr(ctx, X, 4, "X"));
+    CHECK(check_ptr(ctx, pi, 4, "pi"));
+    CHECK(check_ptr(ctx, mu, 4, "mu"));
+    CHECK(check_ptr(ctx, var, 4, "var"));
+    if (!loglik_trace) return fail(ctx, GMM_EINVAL, "loglik_trace is NULL");
+    if (iters < 1) return fail(ctx, GMM_EINVAL, "iters must be >= 1");
+    if (!(var_floor >= 0.f)) return fail(ctx, GMM_EINVAL, "var_floor must be >= 0");
+    if (!(tol >= 0.0)) return fail(ctx, GMM_EINVAL, "tol must be >= 0");
+    DeviceGuard g(ctx->device);
+    int path;
+    CHECK(choose_path(ctx, D, K, &path));
+    CHECK(ensure_scratch(ctx, D, K));
+    const size_t KD = (size_t)K * D;
+    double* Nk = ctx->stats();
+    double* S1 = Nk + K;
+    double* S2 = S1 + KD;
+    int t = 0;
+    for (; t < iters; ++t) {
+        const int slot = t % LL_SLOTS;
+        CHECK(prepare_params(ctx, path, D, K, pi, mu, var));
+        CHECK(zero_stats(ctx, D, K, Nk, S1, S2, slot));
+        CHECK(accumulate_points(ctx, path, X, N, D, K, mu, Nk, S1, S2, slot));
+        KL(launch_finalize(ctx->stream, N, D, K, Nk, S1, S2, var_floor, pi, mu, var));
+        ctx->last_path = path;
+        int rc = read_result(ctx, slot, &loglik_trace[t]);
+        if (rc != GMM_OK) {
+            if (iters_done) *iters_done = t;
+            return rc;
+        }
+        if (tol > 0.0 && t > 0 &&
+            std::fabs(loglik_trace[t] - loglik_trace[t - 1]) <= tol * std::fabs(loglik_trace[t])) {
+            ++t;
+            break;
+        }
+    }
+    if (iters_done) *iters_done = t;
+    return GMM_OK;
+}
+
+int gmm_em_step_host(gmm_ctx* ctx, const float* X_host, int64_t N, int D, int K, const float* pi_host,
+                     const float* mu_host, const float* var_host, double* Nk_host, double* S1_host, double* S2_host,
+                     double* loglik) {
+    CHECK(check_shape(ctx, N, D, K));
+    CHECK(check_ptr(ctx, X_host, 4, "X_host"));
+    CHECK(check_ptr(ctx, pi_host, 4, "pi_host"));
+    CHECK(check_ptr(ctx, mu_host, 4, "mu_host"));
+    CHECK(check_ptr(ctx, var_host, 4, "var_host"));
+    CHECK(check_ptr(ctx, Nk_host, 8, "Nk_host"));
+    CHECK(check_ptr(ctx, S1_host, 8, "S1_host"));
+    CHECK(check_ptr(ctx, S2_host, 8, "S2_host"));
+    if (!loglik) return fail(ctx, GMM_EINVAL, "loglik is NULL");
+    DeviceGuard g(ctx->device);
+    int path;
+    CHECK(choose_path(ctx, D, K, &path));
+    CHECK(ensure_scratch(ctx, D, K));
+    const size_t KD = (size_t)K * D;
+    // one-time resources of the host path
+    if (!ctx->copy_stream) {
+        CU(cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking));
+        for (int b = 0; b < 2; ++b) {
+            CU(cudaEventCreateWithFlags(&ctx->ev_copied[b], cudaEventDisableTiming));
+            CU(cudaEventCreateWithFlags(&ctx->ev_done[b], cudaEventDisableTiming));
+            void* p = nullptr;
+            if (cudaMalloc(&p, STAGE_BYTES) != cudaSuccess) {
+                cudaGetLastError();
+                return fail(ctx, GMM_ENOMEM, "cannot allocate a %zu-byte staging buffer", STAGE_BYTES);
+            }
+            ctx->xstage[b] = static_cast<float*>(p);
+        }
+    }
+    const size_t pfloats = (size_t)K + 2 * KD;
+    if (pfloats > ctx->hparams_floats) {
+        if (ctx->hparams) {
+            CU(cudaStreamSynchronize(ctx->stream));
+            CU(cudaFree(ctx->hparams));
+            ctx->hparams = nullptr;
+        }
+        void* p = nullptr;
+        if (cudaMalloc(&p, pfloats * 4) != cudaSuccess) {
+            cudaGetLastError();
+            return fail(ctx, GMM_ENOMEM, "cannot allocate the parameter copies");
+        }
+        ctx->hparams = static_cast<float*>(p);
+        ctx->hparams_floats = pfloats;
+    }
+    float* pi = ctx->hparams;
+    float* mu = pi + K;
+    float* var = mu + KD;
+    CU(cudaMemcpyAsync(pi, pi_host, (size_t)K * 4, cudaMemcpyHostToDevice, ctx->stream));
+    CU(cudaMemcpyAsync(mu, mu_host, KD * 4, cudaMemcpyHostToDevice, ctx->stream));
+    CU(cudaMemcpyAsync(var, var_host, KD * 4, cudaMemcpyHostToDevice, ctx->stream));
+    double* Nk = ctx->stats();
+    double* S1 = Nk + K;
+    double* S2 = S1 + KD;
+    CHECK(prepare_params(ctx, path, D, K, pi, mu, var));
+    CHECK(zero_stats(ctx, D, K, Nk, S1, S2, 0));
+    const int64_t rows_per_chunk = (int64_t)(STAGE_BYTES / ((size_t)D * 4));
+    if (rows_per_chunk < 1) return fail(ctx, GMM_EINVAL, "D too large for the staging buffer");
+    int c = 0;
+    for (int64_t off = 0; off < N; off += rows_per_chunk, ++c) {
+        const int b = c & 1;
+        const int64_t cnt = (N - off < rows_per_chunk) ? (N - off) : rows_per_chunk;
+        if (c >= 2) CU(cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_done[b], 0));
+        CU(cudaMemcpyAsync(ctx->xstage[b], X_host + off * D, (size_t)cnt * D * 4, cudaMemcpyHostToDevice, ctx->copy_stream));
+        CU(cudaEventRecord(ctx->ev_copied[b], ctx->copy_stream));
+        CU(cudaStreamWaitEvent(ctx->stream, ctx->ev_copied[b], 0));
+        CHECK(accumulate_points(ctx, path, ctx->xstage[b], cnt, D, K, mu, Nk, S1, S2, 0));
+        CU(cudaEventRecord(ctx->ev_done[b], ctx->stream));
+    }
+    CU(cudaMemcpyAsync(Nk_host, Nk, (size_t)K * 8, cudaMemcpyDeviceToHost, ctx->stream));
+    CU(cudaMemcpyAsync(S1_host, S1, KD * 8, cudaMemcpyDeviceToHost, ctx->stream));
+    CU(cudaMemcpyAsync(S2_host, S2, KD * 8, cudaMemcpyDeviceToHost, ctx->stream));
+    ctx->last_path = path;
+    return read_result(ctx, 0, loglik);
+}
+
+int gmm_assign_topm(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const float* pi, const float* mu,
+                    const float* var, int m, int32_t* idx, float* resp) {
+    CHECK(check_shape(ctx, N, D, K));
+    CHECK(check_ptr(ctx, X, 4, "X"));
+    CHECK(check_ptr(ctx, pi, 4, "pi"));
+    CHECK(check_ptr(ctx, mu, 4, "mu"));
+    CHECK(check_ptr(ctx, var, 4, "var"));
+    CHECK(check_ptr(ctx, idx, 4, "idx"));
+    CHECK(check_ptr(ctx, resp, 4, "resp"));
+    if (m < 1 || m > K || m > GMM_MAX_TOPM) return fail(ctx, GMM_EINVAL, "m must be in [1, min(K, %d)] (got %d)", GMM_MAX_TOPM, m);
+    DeviceGuard g(ctx->device);
+    CHECK(ensure_scratch(ctx, D, K));
+    CHECK(prepare_params(ctx, GMM_PATH_FP32, D, K, pi, mu, var));
+    for (int64_t off = 0; off < N; off += SUPER_TILE) {
+        const int64_t cnt = (N - off < SUPER_TILE) ? (N - off) : SUPER_TILE;
+        KL(launch_topm_fp32(ctx->stream, X + off * D, cnt, D, K, mu, ctx->w2(), ctx->c2(), m, idx + off * m, resp + off * m));
+    }
+    ctx->last_path = GMM_PATH_FP32;
+    return GMM_OK;
+}
+
+size_t gmm_scratch_bytes(int D, int K) {
+    if (D < 1 || K < 1) return 0;
+    return scratch_layout(D, K).total;
+}
+
+int64_t gmm_launch_count(const gmm_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int gmm_set_profiling(gmm_ctx* ctx, int on) {
+    if (!ctx) return GMM_EINVAL;
+    ctx->profiling = on != 0;
+    return GMM_OK;
+}
+
+int gmm_kernel_time(gmm_ctx* ctx, double* total_ms, int64_t* launches) {
+    if (!ctx || !total_ms || !launches) return GMM_EINVAL;
+    DeviceGuard g(ctx->device);
+    CU(cudaStreamSynchronize(ctx->stream));
+    for (int i = 0; i < ctx->ev_used; ++i) {
+        float ms = 0.f;
+        CU(cudaEventElapsedTime(&ms, ctx->ev_a[i], ctx->ev_b[i]));
+        ctx->prof_ms += ms;
+    }
+    ctx->ev_used = 0;
+    *total_ms = ctx->prof_ms;
+    *launches = ctx->prof_launches;
+    return GMM_OK;
+}
+
+int gmm_reset_counters(gmm_ctx* ctx) {
+    if (!ctx) return GMM_EINVAL;
+    ctx->launches = 0;
+    ctx->prof_ms = 0.0;
+    ctx->prof_launches = 0;
+    ctx->ev_used = 0;
+    return GMM_OK;
+}
+
+const char* gmm_strerror(int code) {
+    switch (code) {
+        case GMM_OK: return "ok";
+        case GMM_EINVAL: return "invalid argument";
+        case GMM_EALIGN: return "misaligned pointer";
+        case GMM_ENOMEM: return "out of device memory";
+        case GMM_ECUDA: return "CUDA error";
+        case GMM_ENUMERIC: return "numerical error (invalid parameters or non-finite log-likelihood)";
+        case GMM_ETIMEOUT: return "device-side wait timed out";
+        case GMM_EUNSUPPORTED: return "kernel path does not support this shape";
+        default: return "unknown error";
+    }
+}
+
+const char* gmm_last_error(const gmm_ctx* ctx) { return ctx ? ctx->err : "null context"; }
+
+const char* gmm_version(void) { return "flashgmm 0.1 (sm_100a)"; }
+
+}  // extern "C"

@@ -1,0 +1,50 @@
+// Internal declarations of libflashgmm (not part of the C ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stddef.h>
+#include "../../include/flashgmm.h"
+
+namespace fg {
+
+// Points per super-tile of the two-phase FP32 path: log Z_i of one super-tile lives in a fixed-size scratch buffer,
+// so scratch memory is independent of N.
+constexpr int64_t SUPER_TILE = 1 << 20;
+constexpr int FP32_TILE_P = 64;    // points per CTA tile
+constexpr int FP32_TILE_C = 64;    // components per CTA tile
+constexpr int FP32_MSTEP_DC = 128; // dimensions per M-step CTA
+constexpr int FP32_TARGET_CTAS = 296;
+constexpr int LL_SLOTS = 64;       // device slots for log-likelihood values (gmm_fit keeps one per iteration in a ring)
+
+// Status word bits written by device code, read by the host after a synchronising call.
+enum : int { ST_BAD_VAR = 1, ST_BAD_PI = 2, ST_NONFINITE = 4, ST_TIMEOUT = 8 };
+
+struct Fp32Plan {
+    int comp_blocks, d_chunks, splits;
+};
+Fp32Plan fp32_plan(int D, int K);
+size_t fp32_partial_floats(int D, int K);   // floats in the per-CTA partial buffer
+
+// ---- FP32 (CUDA-core) path -----------------------------------------------------------------------------------
+cudaError_t launch_prepare_fp32(cudaStream_t s, int D, int K, const float* pi, const float* mu, const float* var,
+                                float* w2, float* c2, int* status);
+// log2-domain log Z of n points -> logZ2[n]; per-block float64 partial log-likelihoods -> llpart[ceil(n/64)]
+cudaError_t launch_lse_fp32(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu,
+                            const float* w2, const float* c2, float* logZ2, double* llpart);
+cudaError_t launch_mstep_fp32(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu,
+                              const float* w2, const float* c2, const float* logZ2, float* partials,
+                              const Fp32Plan& plan);
+cudaError_t launch_topm_fp32(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu,
+                             const float* w2, const float* c2, int m, int32_t* idx, float* resp);
+
+// ---- shared by all paths -------------------------------------------------------------------------------------
+// stats (+)= sum over `splits` partial blocks, fixed order, float64.  Partial layout: [splits][K + 2*K*D] floats,
+// each block being (N_k [K], S1 [K*D], S2 [K*D]).
+cudaError_t launch_reduce_partials(cudaStream_t s, int D, int K, int splits, const float* partials, double* Nk,
+                                   double* S1, double* S2, bool accumulate);
+// *ll (+)= sum of llpart[0..n) in a fixed order
+cudaError_t launch_reduce_ll(cudaStream_t s, const double* llpart, int64_t n, double* ll, bool accumulate);
+cudaError_t launch_finalize(cudaStream_t s, int64_t N, int D, int K, const double* Nk, const double* S1,
+                            const double* S2, float var_floor, float* pi, float* mu, float* var);
+
+}  // namespace fg

@@ -1,0 +1,76 @@
+// Deterministic cross-CTA reduction of the per-CTA partial statistics, log-likelihood reduction, and the parameter
+// update (paper Algorithm 1: the atomic adds of its line "Atomically add ..." are replaced by per-CTA partials
+// summed in a fixed order in float64; its last line is the finalize kernel, with Eq. 3 taken per dimension).
+#include "internal.cuh"
+
+namespace fg {
+
+namespace {
+
+__global__ void reduce_partials_kernel(int D, int K, int splits, const float* __restrict__ partials,
+                                       double* __restrict__ Nk, double* __restrict__ S1, double* __restrict__ S2,
+                                       int accumulate) {
+    const size_t KD = (size_t)K * D, per = (size_t)K + 2 * KD;
+    const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= per) return;
+    double s = 0.0;
+    for (int p = 0; p < splits; ++p) s += (double)partials[(size_t)p * per + e];      // fixed order
+    double* dst = (e < (size_t)K) ? (Nk + e) : (e < K + KD) ? (S1 + (e - K)) : (S2 + (e - K - KD));
+    *dst = accumulate ? (*dst + s) : s;
+}
+
+// One block; thread t sums elements t, t + 256, ... in order, then a fixed-shape tree adds the 256 partials.
+__global__ void reduce_ll_kernel(const double* __restrict__ llpart, int64_t n, double* __restrict__ ll,
+                                 int accumulate) {
+    __shared__ double red[256];
+    double s = 0.0;
+    for (int64_t i = threadIdx.x; i < n; i += 256) s += llpart[i];
+    red[threadIdx.x] = s;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) {
+        if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) *ll = accumulate ? (*ll + red[0]) : red[0];
+}
+
+__global__ void finalize_kernel(int64_t N, int D, int K, const double* __restrict__ Nk, const double* __restrict__ S1,
+                                const double* __restrict__ S2, float var_floor, float* __restrict__ pi,
+                                float* __restrict__ mu, float* __restrict__ var) {
+    const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= (size_t)K * D) return;
+    const int k = (int)(e / D);
+    const double nk = Nk[k];
+    if (e % D == 0) pi[k] = (float)(nk / (double)N);                      // pi_k = N_k / N
+    if (nk < 1e-12) return;                                               // empty component keeps mu, var
+    const double m = S1[e] / nk;                                          // Eq. 2
+    double v = S2[e] / nk - m * m;                                        // Eq. 3 per dimension, new mean
+    const double fl = (double)var_floor;
+    if (!(v > fl)) v = fl;
+    mu[e] = (float)m;
+    var[e] = (float)v;
+}
+
+}  // namespace
+
+cudaError_t launch_reduce_partials(cudaStream_t s, int D, int K, int splits, const float* partials, double* Nk,
+                                   double* S1, double* S2, bool accumulate) {
+    const size_t per = (size_t)K + 2 * (size_t)K * D;
+    const unsigned blocks = (unsigned)((per + 255) / 256);
+    reduce_partials_kernel<<<blocks, 256, 0, s>>>(D, K, splits, partials, Nk, S1, S2, accumulate ? 1 : 0);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_reduce_ll(cudaStream_t s, const double* llpart, int64_t n, double* ll, bool accumulate) {
+    reduce_ll_kernel<<<1, 256, 0, s>>>(llpart, n, ll, accumulate ? 1 : 0);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_finalize(cudaStream_t s, int64_t N, int D, int K, const double* Nk, const double* S1,
+                            const double* S2, float var_floor, float* pi, float* mu, float* var) {
+    const size_t n = (size_t)K * D;
+    finalize_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(N, D, K, Nk, S1, S2, var_floor, pi, mu, var);
+    return cudaGetLastError();
+}
+
+}  // namespace fg

@@ -83,14 +83,16 @@ def sample_host(spec: MixtureSpec, n: int | None = None, stream: int = 0) -> np.
     return X
 
 
-def sample_device(spec: MixtureSpec, device, n: int | None = None, chunk_rows: int = 1 << 20):
-    """n (default spec.N) points as a float32 torch tensor [n, D] generated on ``device`` in chunks."""
+def sample_device(spec: MixtureSpec, device, n: int | None = None, chunk_rows: int = 1 << 20, stream: int = 0):
+    """n (default spec.N) points as a float32 torch tensor [n, D] generated on ``device`` in chunks.
+
+    ``stream`` selects an independent draw from the same mixture (one per rank in a sharded run)."""
     import torch
 
     n = spec.N if n is None else int(n)
     w, means, stds = true_params(spec)
     gen = torch.Generator(device=device)
-    gen.manual_seed(spec.seed * 1_000_003 + 17)
+    gen.manual_seed(spec.seed * 1_000_003 + 17 + 7919 * stream)
     cdf = torch.tensor(np.cumsum(w), dtype=torch.float64, device=device)
     means_d = torch.tensor(means, dtype=torch.float32, device=device)
     stds_d = torch.tensor(stds, dtype=torch.float32, device=device)

@@ -1,0 +1,309 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the float64 CPU oracle on the same seeded inputs.
+
+Tolerances and the two comparison modes (teacher-forced / free-running) are defined in tests/parity_util.py.
+Every test here runs for each kernel path that supports the shape (FP32 CUDA-core path: any shape; tensor-core
+path: see include/flashgmm.h).
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import gmm_oracle as orc
+from paper_2606_10896_b200 import synth
+from tests.parity_util import assert_params_close, assert_stats_close, assert_topm_matches, data_scale
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module")
+def fg():
+    from paper_2606_10896_b200 import flashgmm
+
+    return flashgmm
+
+
+@pytest.fixture()
+def ctx(fg):
+    c = fg.Context(0)
+    yield c
+    c.close()
+
+
+def _t(a, dtype=torch.float32):
+    return torch.as_tensor(np.ascontiguousarray(a), dtype=dtype, device=DEV).contiguous()
+
+
+def _paths(fg, D, K):
+    paths = [fg.GMM_PATH_FP32]
+    if tensor_path_supports(fg, D, K):
+        paths.append(fg.GMM_PATH_TENSOR)
+    return paths
+
+
+def tensor_path_supports(fg, D, K):
+    probe = getattr(fg, "tensor_path_supports", None)
+    return bool(probe and probe(D, K))
+
+
+def _gpu_step(ctx, X_d, pi, mu, var):
+    Nk, S1, S2, L = ctx.gmm_em_step(X_d, _t(pi), _t(mu), _t(var))
+    return Nk.cpu().numpy(), S1.cpu().numpy(), S2.cpu().numpy(), L
+
+
+def _teacher_forced(fg, ctx, X, spec, iters, paths=None):
+    N, D = X.shape
+    s = data_scale(X)
+    pi0, mu0, var0 = synth.init_params(X, spec)
+    ref = orc.fit(X, pi0, mu0, var0, iters, var_floor=spec.var_floor, keep_params=True)
+    X_d = _t(X)
+    for path in (paths or _paths(fg, D, spec.K)):
+        ctx.gmm_set_path(path)
+        for t in range(iters):
+            p_t, m_t, v_t = ref["params"][t]
+            # the GPU holds float32 parameters: step both sides from the same float32 values
+            p32, m32, v32 = p_t.astype(np.float32), m_t.astype(np.float32), v_t.astype(np.float32)
+            Nk_r, S1_r, S2_r, L_r = orc.em_step(X, p32, m32, v32)
+            pr, mr, vr, _, _, _ = orc.em_iteration(X, p32, m32, v32, var_floor=spec.var_floor)
+            Nk_g, S1_g, S2_g, L_g = _gpu_step(ctx, X_d, p32, m32, v32)
+            what = f"path {path} iteration {t}"
+            assert abs(L_g - L_r) <= 1e-5 * abs(L_r), f"{what}: loglik {L_g} vs {L_r}"
+            assert abs(Nk_g.sum() - N) <= 1e-6 * N * 10, f"{what}: sum N_k = {Nk_g.sum()} vs N = {N}"
+            assert_stats_close(N, s, (Nk_g, S1_g, S2_g), (Nk_r, S1_r, S2_r), what)
+            pi_d, mu_d, var_d = _t(p32), _t(m32), _t(v32)
+            ctx.gmm_finalize(N, _t(Nk_g, torch.float64), _t(S1_g, torch.float64), _t(S2_g, torch.float64),
+                             spec.var_floor, pi_d, mu_d, var_d)
+            assert_params_close(N, s, (pi_d.cpu().numpy(), mu_d.cpu().numpy(), var_d.cpu().numpy()), (pr, mr, vr),
+                                Nk_r, what)
+        assert ctx.gmm_last_path() == path
+
+
+def test_config1_teacher_forced_10_iterations(fg, ctx):
+    spec = synth.CONFIGS[1]
+    _teacher_forced(fg, ctx, synth.sample_host(spec), spec, spec.iters)
+
+
+def test_config1_free_running_fit(fg, ctx):
+    spec = synth.CONFIGS[1]
+    X = synth.sample_host(spec)
+    pi0, mu0, var0 = synth.init_params(X, spec)
+    ref = orc.fit(X, pi0, mu0, var0, spec.iters, var_floor=spec.var_floor)
+    for path in _paths(fg, spec.D, spec.K):
+        ctx.gmm_set_path(path)
+        pi, mu, var = _t(pi0), _t(mu0), _t(var0)
+        trace, done = ctx.gmm_fit(_t(X), pi, mu, var, spec.iters, spec.var_floor)
+        assert done == spec.iters
+        np.testing.assert_allclose(trace, ref["trace"], rtol=1e-4)
+        assert (np.diff(trace) >= -1e-6 * np.abs(trace[1:])).all()
+        s = data_scale(X)
+        Nk = orc.em_step(X, ref["pi"], ref["mu"], ref["var"])[0]
+        # after 10 free-running iterations the parameters have not drifted apart
+        assert np.abs(mu.cpu().numpy() - ref["mu"])[Nk >= 1].max() <= 1e-3 * s
+
+
+def test_config2_cut_teacher_forced(fg, ctx):
+    # K=1024, D=128 with N=3000: 47 point tiles of 64 with a ragged tail of 56
+    spec = synth.CONFIGS[2].with_n(3000)
+    _teacher_forced(fg, ctx, synth.sample_host(spec), spec, 3)
+
+
+def test_config2_free_running_30_iterations(fg, ctx):
+    spec = synth.CONFIGS[2].with_n(20_000)
+    X = synth.sample_host(spec)
+    pi0, mu0, var0 = synth.init_params(X, spec)
+    ref = orc.fit(X, pi0, mu0, var0, 30, var_floor=spec.var_floor)
+    for path in _paths(fg, spec.D, spec.K):
+        ctx.gmm_set_path(path)
+        pi, mu, var = _t(pi0), _t(mu0), _t(var0)
+        trace, done = ctx.gmm_fit(_t(X), pi, mu, var, 30, spec.var_floor)
+        assert done == 30
+        np.testing.assert_allclose(trace, ref["trace"], rtol=1e-4)
+
+
+@pytest.mark.parametrize("N,D,K", [(1, 1, 1), (127, 16, 8), (129, 96, 129), (64, 100, 1), (1000, 3, 65),
+                                    (257, 128, 128), (333, 130, 70)])
+def test_odd_shapes_one_step(fg, ctx, N, D, K):
+    rng = np.random.Generator(np.random.PCG64(N * 1000 + D * 10 + K))
+    mu = rng.normal(0, 2, (K, D))
+    var = rng.uniform(0.3, 2.0, (K, D))
+    pi = rng.dirichlet(np.ones(K))
+    X = (mu[rng.integers(0, K, N)] + rng.standard_normal((N, D))).astype(np.float32)
+    s = max(data_scale(X), 1.0)
+    p32, m32, v32 = pi.astype(np.float32), mu.astype(np.float32), var.astype(np.float32)
+    ref = orc.em_step(X, p32, m32, v32)
+    for path in _paths(fg, D, K):
+        ctx.gmm_set_path(path)
+        got = _gpu_step(ctx, _t(X), p32, m32, v32)
+        assert abs(got[3] - ref[3]) <= 1e-5 * abs(ref[3]) + 1e-6
+        assert_stats_close(N, s, got[:3], ref[:3], f"path {path} shape {(N, D, K)}")
+
+
+def test_runs_are_bit_identical(fg, ctx):
+    spec = synth.CONFIGS[2].with_n(5000)
+    X = synth.sample_host(spec)
+    pi, mu, var = synth.init_params(X, spec)
+    X_d = _t(X)
+    for path in _paths(fg, spec.D, spec.K):
+        ctx.gmm_set_path(path)
+        a = _gpu_step(ctx, X_d, pi, mu, var)
+        b = _gpu_step(ctx, X_d, pi, mu, var)
+        for u, v in zip(a[:3], b[:3]):
+            assert np.array_equal(u, v)
+        assert a[3] == b[3]
+
+
+def test_zero_weight_and_far_components(fg, ctx):
+    rng = np.random.Generator(np.random.PCG64(5))
+    X = np.concatenate([rng.normal(0, 1, (200, 4)), rng.normal(8, 1, (200, 4))]).astype(np.float32)
+    mu = np.array([[0.0] * 4, [8.0] * 4, [1e3] * 4, [4.0] * 4], np.float32)
+    var = np.ones((4, 4), np.float32)
+    pi = np.array([0.5, 0.5, 0.0, 0.0], np.float32)
+    ref = orc.em_step(X, pi, mu, var)
+    for path in _paths(fg, 4, 4):
+        ctx.gmm_set_path(path)
+        Nk, S1, S2, L = _gpu_step(ctx, _t(X), pi, mu, var)
+        assert np.isfinite(L) and abs(L - ref[3]) <= 1e-5 * abs(ref[3])
+        assert Nk[2] == 0.0 and Nk[3] == 0.0
+        assert not np.isnan(S1).any() and not np.isnan(S2).any()
+        # finalize keeps the empty components' mean and variance
+        pi_d, mu_d, var_d = _t(pi), _t(mu), _t(var)
+        ctx.gmm_finalize(len(X), _t(Nk, torch.float64), _t(S1, torch.float64), _t(S2, torch.float64), 1e-6, pi_d,
+                         mu_d, var_d)
+        assert np.array_equal(mu_d.cpu().numpy()[2:], mu[2:]) and np.array_equal(var_d.cpu().numpy()[2:], var[2:])
+        assert pi_d.cpu().numpy()[2] == 0.0
+
+
+def test_variance_floor_is_applied(fg, ctx):
+    X = np.concatenate([np.zeros((50, 2)), np.full((50, 2), 10.0)]).astype(np.float32)
+    mu = np.array([[0.0, 0.0], [10.0, 10.0]], np.float32)
+    var = np.ones((2, 2), np.float32)
+    pi = np.array([0.5, 0.5], np.float32)
+    pi_d, mu_d, var_d = _t(pi), _t(mu), _t(var)
+    trace, _ = ctx.gmm_fit(_t(X), pi_d, mu_d, var_d, 2, 1e-3)
+    np.testing.assert_allclose(var_d.cpu().numpy(), 1e-3, rtol=1e-6)
+    ref = orc.fit(X, pi, mu, var, 2, var_floor=1e-3)
+    np.testing.assert_allclose(trace, ref["trace"], rtol=1e-5)
+
+
+def test_invalid_arguments_and_parameters(fg, ctx):
+    X = _t(np.zeros((10, 4), np.float32))
+    pi, mu, var = _t(np.full(2, 0.5)), _t(np.zeros((2, 4))), _t(np.ones((2, 4)))
+    with pytest.raises(fg.GmmError) as e:
+        ctx.gmm_assign_topm(X, pi, mu, var, 3)
+    assert e.value.code == fg.GMM_EINVAL
+    with pytest.raises(fg.GmmError) as e:
+        ctx.gmm_fit(X, pi, mu, var, 0)
+    assert e.value.code == fg.GMM_EINVAL
+    bad = var.clone()
+    bad[1, 2] = 0.0
+    with pytest.raises(fg.GmmError) as e:
+        ctx.gmm_em_step(X, pi, mu, bad)
+    assert e.value.code == fg.GMM_ENUMERIC
+    negpi = _t(np.array([1.5, -0.5]))
+    with pytest.raises(fg.GmmError) as e:
+        ctx.gmm_em_step(X, negpi, mu, var)
+    assert e.value.code == fg.GMM_ENUMERIC
+    # the context is still usable afterwards
+    ctx.gmm_em_step(X, pi, mu, var)
+    # misaligned pointer
+    buf = torch.zeros(10 * 4 * 4 + 8, dtype=torch.uint8, device=DEV)
+    rc = fg.lib.gmm_em_step(ctx._h, buf.data_ptr() + 1, 10, 4, 2, pi.data_ptr(), mu.data_ptr(), var.data_ptr(),
+                            torch.zeros(2, dtype=torch.float64, device=DEV).data_ptr(),
+                            torch.zeros(8, dtype=torch.float64, device=DEV).data_ptr(),
+                            torch.zeros(8, dtype=torch.float64, device=DEV).data_ptr(),
+                            __import__("ctypes").byref(__import__("ctypes").c_double()))
+    assert rc == fg.GMM_EALIGN
+
+
+def test_host_streaming_matches_device_call(fg, ctx):
+    spec = synth.CONFIGS[2].with_n(4000)
+    X = synth.sample_host(spec)
+    pi, mu, var = synth.init_params(X, spec)
+    for path in _paths(fg, spec.D, spec.K):
+        ctx.gmm_set_path(path)
+        a = _gpu_step(ctx, _t(X), pi, mu, var)
+        b = ctx.gmm_em_step_host(X, pi, mu, var)
+        for u, v in zip(a[:3], b[:3]):
+            assert np.array_equal(u, v)
+        assert a[3] == b[3]
+
+
+def test_host_streaming_multiple_chunks_is_additive(fg, ctx):
+    # D=2048 makes a staging chunk hold 16384 rows, so 40000 rows take three chunks
+    rng = np.random.Generator(np.random.PCG64(77))
+    N, D, K = 40_000, 2048, 4
+    mu = rng.normal(0, 1, (K, D)).astype(np.float32)
+    var = rng.uniform(0.5, 1.5, (K, D)).astype(np.float32)
+    pi = np.full(K, 1 / K, np.float32)
+    X = (mu[rng.integers(0, K, N)] + rng.standard_normal((N, D), dtype=np.float32)).astype(np.float32)
+    ctx.gmm_set_path(fg.GMM_PATH_FP32)
+    a = _gpu_step(ctx, _t(X), pi, mu, var)
+    b = ctx.gmm_em_step_host(X, pi, mu, var)
+    for u, v in zip(a[:3], b[:3]):
+        np.testing.assert_allclose(u, v, rtol=1e-6, atol=1e-6)
+    assert b[3] == pytest.approx(a[3], rel=1e-9)
+
+
+@pytest.mark.parametrize("cfg,n,m", [(1, 2000, 1), (1, 2000, 2), (1, 1999, 4), (1, 500, 8), (2, 1500, 2), (2, 700, 4)])
+def test_topm_against_oracle(fg, ctx, cfg, n, m):
+    spec = synth.CONFIGS[cfg].with_n(n)
+    X = synth.sample_host(spec)
+    pi0, mu0, var0 = synth.init_params(X, spec)
+    fit = orc.fit(X, pi0, mu0, var0, 3, var_floor=spec.var_floor)
+    p32, m32, v32 = (fit[k].astype(np.float32) for k in ("pi", "mu", "var"))
+    idx_r, resp_r, next_r = orc.topm(X, p32, m32, v32, m)
+    idx_g, resp_g = ctx.gmm_assign_topm(_t(X), _t(p32), _t(m32), _t(v32), m)
+    torch.cuda.synchronize()
+    assert_topm_matches(idx_g.cpu().numpy(), resp_g.cpu().numpy(), idx_r, resp_r, next_r, what=f"cfg {cfg} m {m}")
+
+
+def test_topm_exact_ties_go_to_the_smaller_index(fg, ctx):
+    X = _t(np.zeros((70, 4), np.float32))
+    K = 6
+    idx, resp = ctx.gmm_assign_topm(X, _t(np.full(K, 1 / K)), _t(np.zeros((K, 4))), _t(np.ones((K, 4))), 3)
+    torch.cuda.synchronize()
+    assert np.array_equal(idx.cpu().numpy(), np.tile([0, 1, 2], (70, 1)))
+    np.testing.assert_allclose(resp.cpu().numpy(), 1 / K, rtol=1e-5)
+
+
+def test_scratch_does_not_grow_with_n(fg, ctx):
+    assert fg.gmm_scratch_bytes(128, 1024) == fg.gmm_scratch_bytes(128, 1024)
+    spec = synth.CONFIGS[2]
+    Xs = synth.sample_device(spec.with_n(2_000), DEV)
+    Xl = synth.sample_device(spec.with_n(300_000), DEV)
+    pi, mu, var = (_t(a) for a in synth.init_params(Xs, spec.with_n(2_000)))
+    ctx.gmm_em_step(Xs, pi, mu, var)
+    torch.cuda.synchronize()
+    free_small = torch.cuda.mem_get_info()[0]
+    ctx.gmm_em_step(Xl, pi, mu, var)
+    torch.cuda.synchronize()
+    free_large = torch.cuda.mem_get_info()[0]
+    assert free_small == free_large, "device memory in use changed with N"
+
+
+def test_config3_full_size_conservation_and_subsample(fg, ctx):
+    """N = 1M, K = 1024, D = 128 in the launch configuration the benchmark times: conservation laws at full N
+    (sum_k N_k = N, sum_k S1 = column sums of X, sum_k S2 = column sums of X^2) and one oracle step on a seeded
+    50K-row subsample that the GPU re-runs on the same rows."""
+    spec = synth.CONFIGS[3]
+    X = synth.sample_device(spec, DEV)
+    pi0, mu0, var0 = synth.init_params(X, spec)
+    N = spec.N
+    col1 = X.double().sum(0).cpu().numpy()
+    col2 = (X.double() ** 2).sum(0).cpu().numpy()
+    rows = synth.subsample_rows(N, 50_000, spec.seed)
+    Xsub_d = X[torch.as_tensor(rows, device=DEV)].contiguous()
+    Xsub = Xsub_d.cpu().numpy()
+    s = data_scale(Xsub)
+    ref = orc.em_step(Xsub, pi0, mu0, var0)
+    for path in _paths(fg, spec.D, spec.K):
+        ctx.gmm_set_path(path)
+        Nk, S1, S2, L = _gpu_step(ctx, X, pi0, mu0, var0)
+        assert abs(Nk.sum() - N) <= 1e-6 * N
+        np.testing.assert_allclose(S1.sum(0), col1, rtol=1e-5, atol=1e-5 * N * s)
+        np.testing.assert_allclose(S2.sum(0), col2, rtol=1e-5)
+        assert np.isfinite(L)
+        got = _gpu_step(ctx, Xsub_d, pi0, mu0, var0)
+        assert abs(got[3] - ref[3]) <= 1e-5 * abs(ref[3])
+        assert_stats_close(len(rows), s, got[:3], ref[:3], f"path {path} config 3 subsample")

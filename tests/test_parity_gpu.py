@@ -241,7 +241,8 @@ def test_host_streaming_multiple_chunks_is_additive(fg, ctx):
     a = _gpu_step(ctx, _t(X), pi, mu, var)
     b = ctx.gmm_em_step_host(X, pi, mu, var)
     for u, v in zip(a[:3], b[:3]):
-        np.testing.assert_allclose(u, v, rtol=1e-6, atol=1e-6)
+        # float32 per-CTA partials are grouped differently when the points arrive in chunks
+        np.testing.assert_allclose(u, v, rtol=1e-5, atol=1e-5 * np.abs(v).max())
     assert b[3] == pytest.approx(a[3], rel=1e-9)
 
 

@@ -108,6 +108,30 @@ int gmm_assign_topm(gmm_ctx* ctx, const float* X, int64_t N, int D, int K,
                     const float* pi, const float* mu, const float* var, int m,
                     int32_t* idx, float* resp);
 
+/* The statistics of gmm_em_step for callers that cannot allocate device memory.  (The paper has no counterpart of
+ * this entry point; it exists for the library's users.)
+ *
+ * Who needs it: a host that must not call cudaMalloc/cudaFree where it takes an EM step -- a plugin running inside
+ * a service whose device memory is budgeted and owned by another allocator, code called between a framework's own
+ * allocations where a driver allocation would stall the device, or a latency-bound loop that may not block on the
+ * driver's allocator.  This function needs no context and allocates nothing: all scratch of the FP32 kernel chain
+ * lives in a 6 MiB array that is part of the library's device image (every GPU that loads the library holds those
+ * 6 MiB until the process exits).  It calls no cudaMalloc, no cudaFree and no allocating library routine.
+ *
+ *   device, cuda_stream: the device to run on and a cudaStream_t on it (NULL = legacy default stream).
+ *   X, pi, mu, var, Nk, S1, S2: device arrays exactly as for gmm_em_step; loglik: host output.
+ *   Limits: K <= 1024 and K * D <= 32768; larger shapes return GMM_EUNSUPPORTED and launch nothing.
+ *   Always the FP32 path.  Results equal gmm_em_step's up to float32 summation order (the per-CTA partials are
+ *   grouped differently), i.e. well inside the tolerances of the parity tests; they are still deterministic.
+ *   The first call on each device looks up the array's device address (cudaGetSymbolAddress): make that first call
+ *   before starting any stream capture.
+ *   Every call on a device shares the one array and the array keeps the previous call's contents; the function
+ *   clears what it accumulates into, but two calls that overlap on the same GPU (different streams or threads)
+ *   race on it -- serialise them.  Synchronises the stream before returning. */
+int gmm_em_step_static(int device, void* cuda_stream, const float* X, int64_t N, int D, int K,
+                       const float* pi, const float* mu, const float* var,
+                       double* Nk, double* S1, double* S2, double* loglik);
+
 /* Bytes of device scratch a context holds for shape (D, K); independent of N. */
 size_t gmm_scratch_bytes(int D, int K);
 

@@ -44,6 +44,10 @@ EXPORTS = {
     "gmm_assign_topm": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_int,
                                        ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int,
                                        ctypes.c_void_p, ctypes.c_void_p]),
+    "gmm_em_step_static": (ctypes.c_int, [ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int,
+                                          ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                          ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                          ctypes.POINTER(ctypes.c_double)]),
     "gmm_scratch_bytes": (ctypes.c_size_t, [ctypes.c_int, ctypes.c_int]),
     "gmm_launch_count": (ctypes.c_int64, [ctypes.c_void_p]),
     "gmm_set_profiling": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int]),
@@ -94,6 +98,27 @@ def _host(a: np.ndarray, dtype, shape, name: str):
     if not isinstance(a, np.ndarray) or a.dtype != dtype or tuple(a.shape) != tuple(shape) or not a.flags.c_contiguous:
         raise TypeError(f"{name} must be a C-contiguous numpy {np.dtype(dtype).name} array of shape {tuple(shape)}")
     return ctypes.c_void_p(a.ctypes.data)
+
+
+def gmm_em_step_static(X, pi, mu, var, out, stream: torch.cuda.Stream | None = None):
+    """gmm_em_step for callers that may not allocate device memory: no context, scratch in the library's own
+    static device array (K <= 1024, K * D <= 32768).  ``out`` = (Nk, S1, S2) preallocated float64 CUDA tensors --
+    this wrapper allocates nothing on the device either.  Returns the log-likelihood.  Calls that overlap on one
+    GPU race on the shared scratch; the first call on a device should precede any stream capture."""
+    N, D = X.shape
+    K = pi.shape[0]
+    Nk, S1, S2 = out
+    st = stream if stream is not None else torch.cuda.current_stream(X.device)
+    ll = ctypes.c_double(0.0)
+    rc = lib.gmm_em_step_static(X.device.index or 0, ctypes.c_void_p(st.cuda_stream),
+                                _dev(X, torch.float32, (N, D), "X"), N, D, K,
+                                _dev(pi, torch.float32, (K,), "pi"), _dev(mu, torch.float32, (K, D), "mu"),
+                                _dev(var, torch.float32, (K, D), "var"),
+                                _dev(Nk, torch.float64, (K,), "Nk"), _dev(S1, torch.float64, (K, D), "S1"),
+                                _dev(S2, torch.float64, (K, D), "S2"), ctypes.byref(ll))
+    if rc != GMM_OK:
+        raise GmmError(rc, "gmm_em_step_static failed")
+    return ll.value
 
 
 class Context:

@@ -60,6 +60,11 @@ int gmm_destroy(gmm_ctx* ctx);
 /* Select the kernel path for later calls (default GMM_PATH_AUTO).  GMM_EUNSUPPORTED is reported by the compute
  * call, not here, if a forced path cannot run the shape. */
 int gmm_set_path(gmm_ctx* ctx, int path);
+/* 1 if the tensor-core path can run shape (D, K) (D <= 128 and K <= 1024), else 0; GMM_PATH_AUTO uses it whenever
+ * this returns 1.  Components too ill-conditioned for the expanded quadratic form (sum_d mu^2 / var beyond what a
+ * 22-bit split resolves, e.g. a component collapsed onto one point) have their competitive logits recomputed
+ * exactly inside the kernel. */
+int gmm_tensor_path_supports(int D, int K);
 /* The path (GMM_PATH_FP32 or GMM_PATH_TENSOR) the most recent compute call actually ran. */
 int gmm_last_path(const gmm_ctx* ctx);
 

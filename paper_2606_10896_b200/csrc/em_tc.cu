@@ -1,0 +1,894 @@
+// Tensor-core path (sm_100a, tcgen05 + TMEM): the fused E+M tile kernel on the expanded quadratic form.
+//
+// What one launch computes (paper Algorithm 1, both sweeps, for every tile of 64 points):
+//   E-step   L[k, i] = sum_c P[k, c] * Y[i, c]         P = per-component coefficients (a = log2e mu/var, b = -log2e/(2 var)),
+//                                                      Y = [x | x^2], contraction length 2 * 128 padded dimensions
+//   log2 z_ik = t_k * L[k, i] + c_k                     (row scale t_k, constant c_k = log2e (log pi_k - 1/2 sum_d (mu^2/var + log 2 pi var)))
+//   log-sum-exp over ALL K components of a point        (warp butterflies, then one (max, sum) exchange per tile between the CTAs of a cluster
+//                                                        through distributed shared memory: each CTA owns 128 components)
+//   r_ik = 2^(log2 z_ik - log2 Z_i)                     on chip only: written back into TMEM as the A operand of the M-step
+//   M-step   S[k, c] += sum_i r_ik * Y[i, c]            accumulators stationary in TMEM for the CTA's whole life
+// Precision: every operand is split into two fp16 values (hi + lo, 22 bits).  E-step = P_hi Y_hi + P_hi Y_lo + P_lo Y_hi,
+// M-step = r_hi Y_hi + r_hi Y_lo + r_lo Y_hi, fp32 accumulation in TMEM.  Columns of P / Y are interleaved so that one
+// k-step of 16 holds [8 dims of x | the same 8 dims of x^2], which keeps partial sums small.  N_k is summed from the same
+// rounded r (hi + lo) that feeds the M-step.  Accumulators are flushed to float64 partials every TC_FLUSH tiles so that
+// no fp32 accumulation chain is longer than that.
+//
+// Layout: lanes of TMEM = components.  TMEM columns: [0,256) statistics accumulator, [256,384) P_hi (fp16 pairs),
+// [384,448) / [448,512) logits of the two tiles in flight (overwritten in place by r_hi | r_lo).
+// Shared memory: P_lo (64 KB, SW128 K-major), two stages of Y (hi and lo planes, SW128; read K-major by the E-step and
+// MN-major by the M-step), exchange buffers, barriers.
+//
+// Warp roles: warps 0-3 softmax (warp w owns TMEM lanes 32w..32w+31), warps 4-7 load X with coalesced 16-byte loads and
+// build the Y planes, warp 8 issues the MMAs.  Every wait is bounded by a wall-clock limit; on expiry the CTA sets
+// ST_TIMEOUT, all roles leave their loops, TMEM is freed and the kernel returns.
+#include "internal.cuh"
+#include "em_tc.cuh"
+
+#include <cuda_fp16.h>
+#include <math_constants.h>
+
+namespace fg {
+
+namespace {
+
+constexpr int BN = TC_BN;                 // points per tile
+constexpr int NTHREADS = 288;
+constexpr float RSCALE = TC_RSCALE;
+constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
+
+// shared memory map (offsets from a 1024-byte aligned base)
+constexpr int SM_PLO = 0;                       // 65536
+constexpr int SM_Y = 65536;                     // 2 stages x (hi 32768 + lo 32768)
+constexpr int SM_YSTAGE = 65536;
+constexpr int SM_YLO = 32768;
+constexpr int SM_MISC = SM_Y + 2 * SM_YSTAGE;   // 196608
+constexpr int SM_GATHER = SM_MISC;              // 4 warps x 64 floats           1024
+constexpr int SM_WS = SM_GATHER + 1024;         // 4 warps x 64 float2           2048
+constexpr int SM_FAC = SM_WS + 2048;            // 4 warps x 64 floats           1024
+constexpr int SM_EXCH = SM_FAC + 1024;          // 2 bufs x 8 CTAs x 64 float2   8192
+constexpr int SM_SD = SM_EXCH + 8192;           // 128 floats                     512
+constexpr int SM_KAP = SM_SD + 512;             // 128 floats                     512
+constexpr int SM_LL = SM_KAP + 512;             // 64 doubles                     512
+constexpr int SM_BAR = SM_LL + 512;             // barriers                       256
+constexpr int SM_END = SM_BAR + 256;
+constexpr int SMEM_BYTES = SM_END + 1024;       // + alignment slack
+
+enum { B_YFULL0 = 0, B_YFULL1, B_YEMPTY0, B_YEMPTY1, B_LFULL0, B_LFULL1, B_RREADY0, B_RREADY1, B_X0, B_X1, B_ACCFULL,
+       B_ACCFREE, B_FINAL, B_COUNT };
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ unsigned long long gtime() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+__device__ __forceinline__ float fast_ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr >> 4) & 0x3FFF);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
+    d |= (uint64_t)1 << 46;       // descriptor version
+    d |= (uint64_t)2 << 61;       // 128-byte swizzle
+    return d;
+}
+
+__device__ __forceinline__ uint32_t make_idesc(int M, int N, int b_mn_major) {
+    uint32_t d = 0;
+    d |= 1u << 4;                                // D: f32
+    d |= (uint32_t)b_mn_major << 16;             // A, B: f16; A K-major
+    d |= (uint32_t)(N >> 3) << 17;
+    d |= (uint32_t)(M >> 4) << 24;
+    return d;
+}
+
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t acc) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}\n"
+                 ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b, uint32_t idesc, uint32_t acc) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}\n"
+                 ::"r"(d_tmem), "r"(a_tmem), "l"(b), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void mma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ void bar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void bar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void bar_arrive_remote(uint32_t remote_bar) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote_bar) : "memory");
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t cta_rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(cta_rank));
+    return r;
+}
+__device__ __forceinline__ void st_remote_f2(uint32_t remote_addr, float a, float b) {
+    asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(remote_addr), "f"(a), "f"(b) : "memory");
+}
+__device__ __forceinline__ uint32_t cluster_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+// Bounded wait on an mbarrier phase.  Returns false on abort/timeout (and raises the abort flag).
+__device__ __forceinline__ bool bar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, bool cluster_scope) {
+    unsigned long long t0 = 0;
+    for (int it = 0;; ++it) {
+        uint32_t ok;
+        if (cluster_scope)
+            asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
+                         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        else
+            asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
+                         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        if (ok) return true;
+        if (*abort_flag) return false;
+        if ((it & 63) == 63) {
+            const unsigned long long now = gtime();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > WAIT_LIMIT_NS) {
+                *abort_flag = 1;
+                atomicOr(status, ST_TIMEOUT);
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void named_bar_sync(int id, int count) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+
+// ---- TMEM load / store helpers (32 lanes x 32 columns per call; thread = lane) ----
+__device__ __forceinline__ void tmem_ld32(uint32_t addr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+          "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+          "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(addr) : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t addr, const uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+        ::"r"(addr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]),
+          "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]), "r"(v[16]), "r"(v[17]),
+          "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]), "r"(v[24]), "r"(v[25]), "r"(v[26]),
+          "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// ---- warp reduce-scatter butterflies over 64 per-thread values: afterwards lane l holds the reduction (over the
+//      32 lanes) for points 2l and 2l+1.  62 shuffles instead of 64 x 5.
+template <int HALF, bool IS_MAX>
+__device__ __forceinline__ void bfly_round(const float (&v)[2 * HALF], float (&out)[HALF], bool upper, int mask) {
+#pragma unroll
+    for (int j = 0; j < HALF; ++j) {
+        const float mine = upper ? v[HALF + j] : v[j];
+        const float other = upper ? v[j] : v[HALF + j];
+        const float recv = __shfl_xor_sync(0xffffffffu, other, mask);
+        out[j] = IS_MAX ? fmaxf(mine, recv) : (mine + recv);
+    }
+}
+template <bool IS_MAX>
+__device__ __forceinline__ void warp_reduce_scatter(const float (&v)[64], float (&out)[2], int lane) {
+    float a[32], b[16], c[8], d[4];
+    bfly_round<32, IS_MAX>(v, a, lane & 16, 16);
+    bfly_round<16, IS_MAX>(a, b, lane & 8, 8);
+    bfly_round<8, IS_MAX>(b, c, lane & 4, 4);
+    bfly_round<4, IS_MAX>(c, d, lane & 2, 2);
+    bfly_round<2, IS_MAX>(d, out, lane & 1, 1);
+}
+
+__device__ __forceinline__ uint32_t pack_h2(__half lo, __half hi) {
+    return (uint32_t)__half_as_ushort(lo) | ((uint32_t)__half_as_ushort(hi) << 16);
+}
+
+struct TcKernelParams {
+    const float* X;
+    int64_t n;
+    int D, K, CL, Q, n_ks, flush;
+    const uint32_t* phi_img;       // [CL][128 lanes][128] packed fp16 pairs
+    const unsigned char* plo_img;  // [CL][65536] shared-memory image (SW128, K-major)
+    const float* tk;               // [CL*128]
+    const float* ck;               // [CL*128]
+    const float* sd;               // [128] per-dimension power-of-two data scale
+    const float* kap;              // [128] per-dimension shift of the squares: Y = [s x | (s x)^2 + kap]
+    const float* illb;             // [CL*128] 0, or for an ill-conditioned component the log2 margin within which its logits are recomputed exactly
+    const float* mu;               // [K][D] means (exact recomputation)
+    const float* w2;               // [K][D] (log2 e / 2) / var
+    const float* c2;               // [K] log2 e (log pi - 1/2 sum log(2 pi var))
+    double* partial;               // [Q][CL*128][TC_PCOLS]  (+=)
+    double* llpart;                // [Q]
+    int* status;
+#ifdef FLASHGMM_DEBUG
+    float* dbg;      // [Kpad][64] log2 z of the first tile, [Kpad][64] r of the first tile
+#endif
+};
+
+__global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams p) {
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int abort_s;
+    __shared__ int decision_s;
+    volatile int* abort_flag = &abort_s;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t rank = (p.CL > 1) ? cluster_rank() : 0;
+    const int cluster_id = blockIdx.x / p.CL;
+    const int64_t ntiles = (p.n + BN - 1) / BN;
+    const int64_t ntl = (cluster_id < ntiles) ? (ntiles - cluster_id + p.Q - 1) / p.Q : 0;   // tiles of this cluster
+
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SM_BAR);
+    auto BAR = [&](int i) { return smem_u32(&bars[i]); };
+    float* sd_s = reinterpret_cast<float*>(smem + SM_SD);
+    float* kap_s = reinterpret_cast<float*>(smem + SM_KAP);
+
+    if (tid == 0) {
+        abort_s = 0;
+        decision_s = 0;
+        bar_init(BAR(B_YFULL0), 128);  bar_init(BAR(B_YFULL1), 128);
+        bar_init(BAR(B_YEMPTY0), 1);   bar_init(BAR(B_YEMPTY1), 1);
+        bar_init(BAR(B_LFULL0), 1);    bar_init(BAR(B_LFULL1), 1);
+        bar_init(BAR(B_RREADY0), 128); bar_init(BAR(B_RREADY1), 128);
+        bar_init(BAR(B_X0), p.CL * 64); bar_init(BAR(B_X1), p.CL * 64);
+        bar_init(BAR(B_ACCFULL), 1);   bar_init(BAR(B_ACCFREE), 128);
+        bar_init(BAR(B_FINAL), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 8) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(512) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (tid < 128) { sd_s[tid] = p.sd[tid]; kap_s[tid] = p.kap[tid]; }
+    // P_lo image -> shared memory (plain 16-byte copies; the image is already swizzled)
+    {
+        const uint4* src = reinterpret_cast<const uint4*>(p.plo_img + (size_t)rank * 65536);
+        uint4* dst = reinterpret_cast<uint4*>(smem + SM_PLO);
+        for (int i = tid; i < 65536 / 16; i += NTHREADS) dst[i] = __ldg(src + i);
+    }
+    fence_async_smem();
+    fence_before();
+    __syncthreads();
+    fence_after();
+    const uint32_t tmem = tmem_base_s;
+    const uint32_t T_ACC = tmem, T_PHI = tmem + 256, T_LOG = tmem + 384;
+
+    if (warp < 4) {
+        // P_hi -> TMEM (thread = lane = component of this CTA's slice)
+        const uint32_t* src = p.phi_img + ((size_t)rank * 128 + tid) * 128;
+        const uint32_t lane_addr = ((uint32_t)(warp * 32)) << 16;
+#pragma unroll 1
+        for (int c0 = 0; c0 < 128; c0 += 32) {
+            uint32_t v[32];
+#pragma unroll
+            for (int j = 0; j < 32; j += 4) {
+                const uint4 q = __ldg(reinterpret_cast<const uint4*>(src + c0 + j));
+                v[j] = q.x; v[j + 1] = q.y; v[j + 2] = q.z; v[j + 3] = q.w;
+            }
+            tmem_st32(T_PHI + lane_addr + c0, v);
+        }
+        tmem_wait_st();
+    }
+    fence_before();
+    __syncthreads();
+    fence_after();
+    if (p.CL > 1) cluster_sync_all();      // peers' barriers are initialised before anyone sends to them
+
+    if (warp < 4) {
+        // =========================== softmax warps ===========================
+        const uint32_t lane_addr = ((uint32_t)(warp * 32)) << 16;
+        const int kloc = tid;                                   // component within the slice
+        const float tk = p.tk[rank * 128 + kloc];
+        const float ck = p.ck[rank * 128 + kloc];
+        const float illb = p.illb[rank * 128 + kloc];
+        float* gather = reinterpret_cast<float*>(smem + SM_GATHER) + warp * 64;
+        float2* ws = reinterpret_cast<float2*>(smem + SM_WS);          // [4][64]
+        float* fac = reinterpret_cast<float*>(smem + SM_FAC);          // [4][64]
+        float2* exch = reinterpret_cast<float2*>(smem + SM_EXCH);      // [2][8][64]
+        float nk_acc = 0.f;
+        double ll_acc = 0.0;
+        double* prow = p.partial + ((size_t)cluster_id * (p.CL * 128) + rank * 128 + kloc) * TC_PCOLS;
+        uint32_t accfull_parity = 0;
+        bool alive = true;
+
+        // Softmax threads leave the loop only at the uniform decision point after named barrier 2: a thread that
+        // left earlier would strand the others in a hardware barrier.
+        for (int64_t i = 0; i < ntl; ++i) {
+            const int s = (int)(i & 1);
+            const uint32_t ph = (uint32_t)((i >> 1) & 1);
+            const int64_t tile = cluster_id + i * p.Q;
+            const int64_t row0 = tile * BN;
+            const int nvalid = (int)((p.n - row0 < BN) ? (p.n - row0) : BN);
+
+            if (!bar_wait(BAR(B_LFULL0 + s), ph, abort_flag, p.status, false)) alive = false;
+            fence_after();
+            float l[64];
+            {
+                uint32_t v0[32], v1[32];
+                tmem_ld32(T_LOG + s * 64 + lane_addr, v0);
+                tmem_ld32(T_LOG + s * 64 + lane_addr + 32, v1);
+                tmem_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    l[j] = fmaf(__uint_as_float(v0[j]), tk, ck);
+                    l[32 + j] = fmaf(__uint_as_float(v1[j]), tk, ck);
+                }
+            }
+#ifdef FLASHGMM_DEBUG
+            if (p.dbg && cluster_id == 0 && i == 0)
+                for (int j = 0; j < 64; ++j) p.dbg[(size_t)(rank * 128 + kloc) * 64 + j] = l[j];
+#endif
+            // warp-level max per point, all-gathered through shared memory
+            float red[2];
+            warp_reduce_scatter<true>(l, red, lane);
+            reinterpret_cast<float2*>(gather)[lane] = make_float2(red[0], red[1]);
+            __syncwarp();
+            // Ill-conditioned components (sum_d mu^2 / var too large for the 22-bit expanded form, e.g. a component
+            // that collapsed onto a few points): wherever such a component is within reach of the warp's maximum for a
+            // point, its logit is recomputed exactly with direct differences in fp32, the whole warp working on one
+            // (component, point) pair at a time.  Rare by construction: a tight component is competitive for few points.
+            if (__any_sync(0xffffffffu, illb > 0.f)) {
+                uint32_t mlo = 0, mhi = 0;
+                if (illb > 0.f) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        if (j < nvalid && l[j] >= gather[j] - illb) mlo |= 1u << j;
+                        if (32 + j < nvalid && l[32 + j] >= gather[32 + j] - illb) mhi |= 1u << j;
+                    }
+                }
+                bool fixed_any = false;
+                const int kglob = (int)rank * 128 + kloc;
+                for (;;) {
+                    const uint32_t ballot = __ballot_sync(0xffffffffu, (mlo | mhi) != 0u);
+                    if (ballot == 0u) break;
+                    const int src = __ffs(ballot) - 1;
+                    int j = mlo ? (__ffs(mlo) - 1) : (32 + __ffs(mhi) - 1);
+                    j = __shfl_sync(0xffffffffu, j, src);
+                    const int kk = __shfl_sync(0xffffffffu, kglob, src);
+                    const float* xr = p.X + (row0 + j) * p.D;
+                    const float* mr = p.mu + (size_t)kk * p.D;
+                    const float* wr = p.w2 + (size_t)kk * p.D;
+                    float q = 0.f;
+                    for (int d = lane; d < p.D; d += 32) {
+                        const float diff = __ldg(xr + d) - __ldg(mr + d);
+                        q = fmaf(diff * diff, __ldg(wr + d), q);
+                    }
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
+                    const float val = __ldg(p.c2 + kk) - q;
+                    if (lane == src) {
+#pragma unroll
+                        for (int jj = 0; jj < 64; ++jj)
+                            if (jj == j) l[jj] = val;
+                        if (j < 32) mlo &= ~(1u << j); else mhi &= ~(1u << (j - 32));
+                    }
+                    fixed_any = true;
+                }
+                if (fixed_any) {
+                    __syncwarp();
+                    warp_reduce_scatter<true>(l, red, lane);
+                    reinterpret_cast<float2*>(gather)[lane] = make_float2(red[0], red[1]);
+                    __syncwarp();
+                }
+            }
+            const float mw_mine0 = red[0], mw_mine1 = red[1];
+#pragma unroll
+            for (int j = 0; j < 64; j += 4) {
+                const float4 m4 = *reinterpret_cast<const float4*>(gather + j);
+                const float m0 = (m4.x == -CUDART_INF_F) ? 0.f : m4.x;
+                const float m1 = (m4.y == -CUDART_INF_F) ? 0.f : m4.y;
+                const float m2 = (m4.z == -CUDART_INF_F) ? 0.f : m4.z;
+                const float m3 = (m4.w == -CUDART_INF_F) ? 0.f : m4.w;
+                l[j] = fast_ex2(l[j] - m0);
+                l[j + 1] = fast_ex2(l[j + 1] - m1);
+                l[j + 2] = fast_ex2(l[j + 2] - m2);
+                l[j + 3] = fast_ex2(l[j + 3] - m3);
+            }
+            __syncwarp();
+            float sred[2];
+            warp_reduce_scatter<false>(l, sred, lane);
+            *reinterpret_cast<float4*>(&ws[warp * 64 + 2 * lane]) = make_float4(mw_mine0, sred[0], mw_mine1, sred[1]);
+            named_bar_sync(1, 128);
+            if (tid < 64) {
+                const int pt = tid;
+                float2 w4[4];
+#pragma unroll
+                for (int w = 0; w < 4; ++w) w4[w] = ws[w * 64 + pt];
+                float mc = fmaxf(fmaxf(w4[0].x, w4[1].x), fmaxf(w4[2].x, w4[3].x));
+                const float mc_safe = (mc == -CUDART_INF_F) ? 0.f : mc;
+                float sc = 0.f;
+#pragma unroll
+                for (int w = 0; w < 4; ++w)       // a warp whose lanes are all padded / zero-weight has m_w = -inf: skip it
+                    sc += (w4[w].x == -CUDART_INF_F) ? 0.f : w4[w].y * fast_ex2(w4[w].x - mc_safe);
+                // send (m, s) of this CTA's 128 components to every CTA of the cluster (including this one)
+                const uint32_t slot = smem_u32(&exch[(s * 8 + rank) * 64 + pt]);
+                for (int c = 0; c < p.CL; ++c) {
+                    st_remote_f2(map_to_cta(slot, c), mc, sc);
+                    bar_arrive_remote(map_to_cta(BAR(B_X0 + s), c));
+                }
+                if (!bar_wait(BAR(B_X0 + s), ph, abort_flag, p.status, true)) alive = false;
+                float mi = -CUDART_INF_F;
+                float2 e[8];
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    e[c] = (c < p.CL) ? exch[(s * 8 + c) * 64 + pt] : make_float2(-CUDART_INF_F, 0.f);
+                    mi = fmaxf(mi, e[c].x);
+                }
+                const float mi_safe = (mi == -CUDART_INF_F) ? 0.f : mi;
+                float Z = 0.f;
+#pragma unroll
+                for (int c = 0; c < 8; ++c)
+                    Z += (e[c].x == -CUDART_INF_F) ? 0.f : e[c].y * fast_ex2(e[c].x - mi_safe);
+                const bool valid = pt < nvalid;
+                const float inv = (valid && Z > 0.f) ? (RSCALE / Z) : 0.f;
+#pragma unroll
+                for (int w = 0; w < 4; ++w)
+                    fac[w * 64 + pt] = (w4[w].x == -CUDART_INF_F) ? 0.f : fast_ex2(w4[w].x - mi_safe) * inv;
+                if (rank == 0 && valid) ll_acc += (double)(mi + log2f(Z));
+            }
+            if (tid == 0) decision_s = *abort_flag;
+            named_bar_sync(2, 128);
+            if (decision_s) break;
+            // responsibilities: r = p * fac, split into fp16 hi + lo, written over the logits as the M-step A operand
+            {
+                uint32_t hi[32], lo[32];
+                const float* fw = fac + warp * 64;
+                float nsum = 0.f;
+#pragma unroll
+                for (int j = 0; j < 64; j += 4) {
+                    const float4 f4 = *reinterpret_cast<const float4*>(fw + j);
+                    const float r0 = l[j] * f4.x, r1 = l[j + 1] * f4.y, r2 = l[j + 2] * f4.z, r3 = l[j + 3] * f4.w;
+                    const __half h0 = __float2half_rn(r0), h1 = __float2half_rn(r1), h2 = __float2half_rn(r2), h3 = __float2half_rn(r3);
+                    const float b0 = __half2float(h0), b1 = __half2float(h1), b2 = __half2float(h2), b3 = __half2float(h3);
+                    const __half g0 = __float2half_rn(r0 - b0), g1 = __float2half_rn(r1 - b1), g2 = __float2half_rn(r2 - b2), g3 = __float2half_rn(r3 - b3);
+                    nsum += (b0 + __half2float(g0)) + (b1 + __half2float(g1)) + (b2 + __half2float(g2)) + (b3 + __half2float(g3));
+                    hi[j / 2] = pack_h2(h0, h1);
+                    hi[j / 2 + 1] = pack_h2(h2, h3);
+                    lo[j / 2] = pack_h2(g0, g1);
+                    lo[j / 2 + 1] = pack_h2(g2, g3);
+                }
+                nk_acc += nsum;
+                tmem_st32(T_LOG + s * 64 + lane_addr, hi);
+                tmem_st32(T_LOG + s * 64 + lane_addr + 32, lo);
+                tmem_wait_st();
+            }
+            fence_before();
+            bar_arrive(BAR(B_RREADY0 + s));
+
+            // periodic flush of the TMEM accumulators into float64 partials (after the second tile of a pair)
+            const bool pair_end = (i & 1) || (i + 1 == ntl);
+            const int64_t pair_next = (i | 1) + 1;
+            if (pair_end && ((pair_next % p.flush) == 0 || pair_next >= ntl)) {
+                if (!bar_wait(BAR(B_ACCFULL), accfull_parity, abort_flag, p.status, false)) alive = false;
+                accfull_parity ^= 1;
+                fence_after();
+#pragma unroll 1
+                for (int c0 = 0; c0 < 256; c0 += 32) {
+                    uint32_t v[32];
+                    tmem_ld32(T_ACC + lane_addr + c0, v);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) prow[c0 + j] += (double)__uint_as_float(v[j]);
+                }
+                prow[256] += (double)nk_acc;
+                nk_acc = 0.f;
+                fence_before();
+                bar_arrive(BAR(B_ACCFREE));
+            }
+        }
+        if (rank == 0) {
+            double* lls = reinterpret_cast<double*>(smem + SM_LL);
+            if (tid < 64) lls[tid] = ll_acc;
+            named_bar_sync(3, 128);
+            if (tid == 0) {
+                double sum = 0.0;
+                for (int j = 0; j < 64; ++j) sum += lls[j];
+                p.llpart[cluster_id] = sum * 0.69314718055994530942;
+            }
+        }
+    } else if (warp < 8) {
+        // =========================== transform warps: X -> Y planes ===========================
+        const int tau = tid - 128;
+        const int pt = tau >> 1, half = tau & 1;
+        const bool vec_ok = (p.D % 4 == 0) && ((reinterpret_cast<uintptr_t>(p.X) & 15) == 0);
+        for (int64_t i = 0; i < ntl; ++i) {
+            const int s = (int)(i & 1);
+            const uint32_t ph = (uint32_t)((i >> 1) & 1);
+            const int64_t row = (cluster_id + i * p.Q) * BN + pt;
+            const bool row_ok = row < p.n;
+            const float* xr = p.X + row * p.D;
+            if (i >= 2) {
+                if (!bar_wait(BAR(B_YEMPTY0 + s), ph ^ 1, abort_flag, p.status, false)) break;
+            }
+            unsigned char* yhi = smem + SM_Y + s * SM_YSTAGE;
+            unsigned char* ylo = yhi + SM_YLO;
+#pragma unroll 2
+            for (int g = 0; g < 8; ++g) {
+                const int ks = half * 8 + g;
+                const int d0 = ks * 8;
+                float x[8];
+                if (row_ok && vec_ok && d0 + 8 <= p.D) {
+                    const float4 a = __ldg(reinterpret_cast<const float4*>(xr + d0));
+                    const float4 b = __ldg(reinterpret_cast<const float4*>(xr + d0 + 4));
+                    x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) x[j] = (row_ok && d0 + j < p.D) ? __ldg(xr + d0 + j) : 0.f;
+                }
+                uint32_t xh[4], xl[4], qh[4], ql[4];
+#pragma unroll
+                for (int j = 0; j < 8; j += 2) {
+                    float u0 = x[j] * sd_s[d0 + j], u1 = x[j + 1] * sd_s[d0 + j + 1];
+                    u0 = fminf(fmaxf(u0, -240.f), 240.f);
+                    u1 = fminf(fmaxf(u1, -240.f), 240.f);
+                    const float q0 = fmaf(u0, u0, kap_s[d0 + j]), q1 = fmaf(u1, u1, kap_s[d0 + j + 1]);
+                    const __half h0 = __float2half_rn(u0), h1 = __float2half_rn(u1);
+                    const __half g0 = __float2half_rn(u0 - __half2float(h0)), g1 = __float2half_rn(u1 - __half2float(h1));
+                    const __half s0 = __float2half_rn(q0), s1 = __float2half_rn(q1);
+                    const __half t0 = __float2half_rn(q0 - __half2float(s0)), t1 = __float2half_rn(q1 - __half2float(s1));
+                    xh[j / 2] = pack_h2(h0, h1);
+                    xl[j / 2] = pack_h2(g0, g1);
+                    qh[j / 2] = pack_h2(s0, s1);
+                    ql[j / 2] = pack_h2(t0, t1);
+                }
+                // 16-byte chunk index in the point's 512-byte row: 2 ks (x) and 2 ks + 1 (x^2)
+                const int atom = ks >> 2;
+                const int cx = ((2 * (ks & 3)) ^ (pt & 7)) << 4;
+                const int cq = ((2 * (ks & 3) + 1) ^ (pt & 7)) << 4;
+                const int base = atom * 8192 + pt * 128;
+                *reinterpret_cast<uint4*>(yhi + base + cx) = make_uint4(xh[0], xh[1], xh[2], xh[3]);
+                *reinterpret_cast<uint4*>(yhi + base + cq) = make_uint4(qh[0], qh[1], qh[2], qh[3]);
+                *reinterpret_cast<uint4*>(ylo + base + cx) = make_uint4(xl[0], xl[1], xl[2], xl[3]);
+                *reinterpret_cast<uint4*>(ylo + base + cq) = make_uint4(ql[0], ql[1], ql[2], ql[3]);
+            }
+            fence_async_smem();
+            bar_arrive(BAR(B_YFULL0 + s));
+        }
+    } else if (lane == 0) {
+        // =========================== MMA issuer (one thread) ===========================
+        const uint32_t id_e = make_idesc(128, BN, 0);
+        const uint32_t id_m = make_idesc(128, p.n_ks * 16, 1);
+        const uint32_t plo = smem_u32(smem + SM_PLO);
+        bool acc_valid = false;
+        uint32_t accfree_parity = 0;
+        bool alive = true;
+        auto issue_E = [&](int64_t i) -> bool {
+            const int s = (int)(i & 1);
+            const uint32_t ph = (uint32_t)((i >> 1) & 1);
+            if (!bar_wait(BAR(B_YFULL0 + s), ph, abort_flag, p.status, false)) return false;
+            fence_after();
+            const uint32_t yhi = smem_u32(smem + SM_Y + s * SM_YSTAGE), ylo = yhi + SM_YLO;
+            const uint32_t d = T_LOG + s * 64;
+            for (int ks = 0; ks < p.n_ks; ++ks)
+                mma_ts(d, T_PHI + ks * 8, make_desc(yhi + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024), id_e, ks > 0);
+            for (int ks = 0; ks < p.n_ks; ++ks)
+                mma_ts(d, T_PHI + ks * 8, make_desc(ylo + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024), id_e, 1);
+            for (int ks = 0; ks < p.n_ks; ++ks)
+                mma_ss(d, make_desc(plo + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024),
+                       make_desc(yhi + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024), id_e, 1);
+            mma_commit(BAR(B_LFULL0 + s));
+            return true;
+        };
+        auto issue_M = [&](int64_t i) -> bool {
+            const int s = (int)(i & 1);
+            const uint32_t ph = (uint32_t)((i >> 1) & 1);
+            if (!bar_wait(BAR(B_RREADY0 + s), ph, abort_flag, p.status, false)) return false;
+            fence_after();
+            const uint32_t yhi = smem_u32(smem + SM_Y + s * SM_YSTAGE), ylo = yhi + SM_YLO;
+            const uint32_t rhi = T_LOG + s * 64, rlo = rhi + 32;
+            for (int ks = 0; ks < BN / 16; ++ks) {
+                mma_ts(T_ACC, rhi + ks * 8, make_desc(yhi + ks * 2048, 8192, 1024), id_m, acc_valid || ks > 0);
+            }
+            acc_valid = true;
+            for (int ks = 0; ks < BN / 16; ++ks) mma_ts(T_ACC, rhi + ks * 8, make_desc(ylo + ks * 2048, 8192, 1024), id_m, 1);
+            for (int ks = 0; ks < BN / 16; ++ks) mma_ts(T_ACC, rlo + ks * 8, make_desc(yhi + ks * 2048, 8192, 1024), id_m, 1);
+            mma_commit(BAR(B_YEMPTY0 + s));
+            return true;
+        };
+        for (int64_t i = 0; i < ntl && alive; i += 2) {
+            const bool has2 = i + 1 < ntl;
+            alive = issue_E(i);
+            if (alive && has2) alive = issue_E(i + 1);
+            if (alive) alive = issue_M(i);
+            if (alive && has2) alive = issue_M(i + 1);
+            if (!alive) break;
+            const int64_t pair_next = i + 2;
+            if ((pair_next % p.flush) == 0 || pair_next >= ntl) {
+                mma_commit(BAR(B_ACCFULL));
+                if (!bar_wait(BAR(B_ACCFREE), accfree_parity, abort_flag, p.status, false)) { alive = false; break; }
+                accfree_parity ^= 1;
+                fence_after();
+                acc_valid = false;
+            }
+        }
+        // drain: every MMA issued by this thread has completed before TMEM is released
+        mma_commit(BAR(B_FINAL));
+        bar_wait(BAR(B_FINAL), 0, abort_flag, p.status, false);
+    }
+
+    // teardown: everybody meets, peers are done with this CTA's shared memory, TMEM is released
+    fence_before();
+    __syncthreads();
+    if (p.CL > 1) cluster_sync_all();
+    if (warp == 8) {
+        fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------------------
+// Parameter preparation for the tensor path (float64 arithmetic, K*D elements: negligible)
+
+// s_d = 2^-round(log2 rms_d) with rms_d^2 = sum_k pi_k (mu_kd^2 + var_kd): brings every dimension to O(1) so that the
+// fp16 splits keep their precision whatever the data's units.  kap_d = s_d^2 sum_k pi_k mu_kd^2: the squares enter the
+// contraction as (s x)^2 + kap_d, which turns the monotonically growing partial sums sum_d w (mu x - x^2 / 2) ~ sum_d w mu^2 / 2
+// into a zero-mean walk sum_d w (mu^2 - kap) / 2 (several times smaller), and with it the error of the fp32 accumulation
+// in the tensor core.  The constant is given back exactly through c_k (E-step) and kap_d N_k (M-step).
+__global__ void tc_scale_kernel(int D, int K, const float* __restrict__ pi, const float* __restrict__ mu,
+                                const float* __restrict__ var, float* __restrict__ sd, float* __restrict__ kap) {
+    const int d = threadIdx.x;
+    float s = 1.f, kp = 0.f;
+    if (d < D) {
+        double acc = 0.0, accm = 0.0, wsum = 0.0;
+        for (int k = 0; k < K; ++k) {
+            const double w = (double)pi[k];
+            const double m = (double)mu[(size_t)k * D + d];
+            acc += w * (m * m + (double)var[(size_t)k * D + d]);
+            accm += w * m * m;
+            wsum += w;
+        }
+        if (wsum > 0.0) { acc /= wsum; accm /= wsum; }
+        if (acc > 0.0 && isfinite(acc)) {
+            const double e = rint(0.5 * log2(acc));
+            s = (float)exp2(-fmin(fmax(e, -60.0), 60.0));
+            kp = (float)(accm * (double)s * (double)s);      // mean of mu^2 in scaled units
+        }
+    }
+    sd[d] = s;
+    kap[d] = kp;
+}
+
+// One block (128 threads) per padded component: builds the P_hi TMEM image, the P_lo shared-memory image, t_k, c_k,
+// and flags ill-conditioned components.
+__global__ void __launch_bounds__(128) tc_prepare_kernel(int D, int K, const float* __restrict__ pi,
+                                                         const float* __restrict__ mu, const float* __restrict__ var,
+                                                         const float* __restrict__ sd, const float* __restrict__ kap,
+                                                         uint32_t* __restrict__ phi_img,
+                                                         unsigned char* __restrict__ plo_img, float* __restrict__ tk,
+                                                         float* __restrict__ ck, float* __restrict__ illb, float cond_limit,
+                                                         int* __restrict__ status) {
+    const int k = blockIdx.x, d = threadIdx.x;
+    const int slice = k >> 7, row = k & 127;
+    __shared__ double red_max[128], red_c[128], red_cond[128], red_k[128];
+    __shared__ __half hi_s[256], lo_s[256];
+    double a = 0.0, b = 0.0, cterm = 0.0, cond = 0.0;
+    const bool live = (k < K) && (d < D);
+    if (live) {
+        const double v = (double)var[(size_t)k * D + d], m = (double)mu[(size_t)k * D + d], s = (double)sd[d];
+        const double w = 1.4426950408889634074 / v;
+        a = w * m / s;
+        b = -0.5 * w / (s * s);
+        cterm = m * m / v + log(6.283185307179586476925286766559 * v);
+        cond = 0.5 * w * 3.0 * (m * m + 9.0 * v);
+    }
+    red_max[d] = fmax(fabs(a), fabs(b));
+    red_c[d] = cterm;
+    red_cond[d] = cond;
+    __syncthreads();
+    for (int o = 64; o > 0; o >>= 1) {
+        if (d < o) {
+            red_max[d] = fmax(red_max[d], red_max[d + o]);
+            red_c[d] += red_c[d + o];
+            red_cond[d] += red_cond[d + o];
+        }
+        __syncthreads();
+    }
+    const double mx = red_max[0];
+    double t = 1.0;
+    if (mx > 0.0 && isfinite(mx)) t = exp2(floor(log2(mx)) - 9.0);      // max |P / t| in [512, 1024)
+    const double as = a / t, bs = b / t;
+    const __half ah = __double2half(as), bh = __double2half(bs);
+    const __half al = __double2half(as - (double)__half2float(ah)), bl = __double2half(bs - (double)__half2float(bh));
+    // interleaved column order: k-step ks = d / 8 holds [x(8 dims) | x^2(8 dims)]
+    const int cx = 16 * (d >> 3) + (d & 7), cq = cx + 8;
+    hi_s[cx] = ah; hi_s[cq] = bh; lo_s[cx] = al; lo_s[cq] = bl;
+    // what the contraction adds through the shifted squares: t * (b_hi + b_lo) * kap, summed over d, is taken out of c_k
+    red_k[d] = live ? t * ((double)__half2float(bh) + (double)__half2float(bl)) * (double)kap[d] : 0.0;
+    __syncthreads();
+    for (int o = 64; o > 0; o >>= 1) {
+        if (d < o) red_k[d] += red_k[d + o];
+        __syncthreads();
+    }
+    // P_hi image: [slice][row][128] packed pairs (even column in the low half)
+    phi_img[((size_t)slice * 128 + row) * 128 + d] =
+        (uint32_t)__half_as_ushort(hi_s[2 * d]) | ((uint32_t)__half_as_ushort(hi_s[2 * d + 1]) << 16);
+    // P_lo image: SW128 K-major, atoms of 64 columns, 128 rows
+    for (int c = d; c < 256; c += 128) {
+        const int atom = c >> 6, cc = c & 63;
+        const size_t off = (size_t)slice * 65536 + atom * 16384 + row * 128 + ((((cc >> 3) ^ (row & 7)) << 4) | ((cc & 7) << 1));
+        *reinterpret_cast<__half*>(plo_img + off) = lo_s[c];
+    }
+    if (d == 0) {
+        float c = -CUDART_INF_F;
+        if (k < K) {
+            const float pk = pi[k];
+            if (pk > 0.f) c = (float)(1.4426950408889634074 * (log((double)pk) - 0.5 * red_c[0]) - red_k[0]);
+        }
+        tk[k] = (float)t;
+        ck[k] = c;
+        // conditioning estimate of the expanded form: 2^-22 sum_d w2 * 3 (mu^2 + 9 var) ~ absolute log2 error bound
+        const double cond = red_cond[0] * 2.384185791015625e-07;
+        float margin = 0.f;
+        if (k < K && cond > (double)cond_limit) {
+            margin = (float)fmin(40.0 + 8.0 * cond, 1e30);
+            atomicOr(status, ST_ILLCOND);
+        }
+        illb[k] = margin;
+    }
+}
+
+// stats (+)= sum over Q cluster partials (float64, fixed order), undoing the responsibility scale, the per-dimension
+// data scale and the interleaved column order.
+__global__ void tc_reduce_kernel(int D, int K, int Kpad, int Q, const double* __restrict__ partial,
+                                 const float* __restrict__ sd, const float* __restrict__ kap, double* __restrict__ Nk,
+                                 double* __restrict__ S1, double* __restrict__ S2, int accumulate) {
+    const size_t KD = (size_t)K * D, per = (size_t)K + 2 * KD;
+    const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= per) return;
+    int k, col;
+    double unscale = 1.0 / (double)TC_RSCALE;
+    double* dst;
+    if (e < (size_t)K) {
+        k = (int)e; col = 256; dst = Nk + e;
+    } else if (e < K + KD) {
+        const size_t j = e - K; k = (int)(j / D); const int d = (int)(j % D);
+        col = 16 * (d >> 3) + (d & 7); unscale /= (double)sd[d]; dst = S1 + j;
+    } else {
+        const size_t j = e - K - KD; k = (int)(j / D); const int d = (int)(j % D);
+        col = 16 * (d >> 3) + (d & 7) + 8; unscale /= (double)sd[d] * (double)sd[d]; dst = S2 + j;
+    }
+    double s = 0.0;
+    for (int q = 0; q < Q; ++q) s += partial[((size_t)q * Kpad + k) * TC_PCOLS + col];
+    if (e >= K + KD) {          // squares were accumulated as (s x)^2 + kap: take kap * N_k out again
+        const int d = (int)((e - K - KD) % D);
+        double nk = 0.0;
+        for (int q = 0; q < Q; ++q) nk += partial[((size_t)q * Kpad + k) * TC_PCOLS + 256];
+        s -= (double)kap[d] * nk;
+    }
+    s *= unscale;
+    *dst = accumulate ? (*dst + s) : s;
+}
+
+}  // namespace
+
+#ifdef FLASHGMM_DEBUG
+float* g_tc_debug = nullptr;
+extern "C" void gmm_debug_set_buffer(float* p) { g_tc_debug = p; }
+#endif
+
+bool tc_supports(int D, int K) { return D >= 1 && D <= 128 && K >= 1 && K <= 1024; }
+
+TcPlan tc_plan(int D, int K, int num_sms) {
+    TcPlan pl;
+    pl.CL = (K + 127) / 128;
+    pl.Kpad = pl.CL * 128;
+    pl.Q = num_sms / pl.CL;
+    if (pl.Q < 1) pl.Q = 1;
+    pl.n_ks = (D + 7) / 8;
+    return pl;
+}
+
+size_t tc_scratch_bytes(int D, int K) {
+    if (!tc_supports(D, K)) return 0;
+    const TcPlan pl = tc_plan(D, K, 160);
+    size_t b = 0;
+    b += (size_t)pl.CL * 128 * 128 * 4;                    // P_hi image
+    b += (size_t)pl.CL * 65536;                            // P_lo image
+    b += (size_t)pl.Kpad * 4 * 2 + 512;                    // t_k, c_k, s_d
+    b += (size_t)pl.Q * pl.Kpad * TC_PCOLS * 8;            // float64 partials
+    b += (size_t)pl.Q * 8;
+    return b + 8 * 256;
+}
+
+cudaError_t launch_prepare_tc(cudaStream_t s, int D, int K, const float* pi, const float* mu, const float* var,
+                              const TcBuffers& tb, float cond_limit, int* status) {
+    const TcPlan pl = tc_plan(D, K, 148);
+    tc_scale_kernel<<<1, 128, 0, s>>>(D, K, pi, mu, var, tb.sd, tb.kap);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    tc_prepare_kernel<<<pl.Kpad, 128, 0, s>>>(D, K, pi, mu, var, tb.sd, tb.kap, tb.phi_img, tb.plo_img, tb.tk, tb.ck, tb.illb, cond_limit, status);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_em_tc(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu, const float* w2,
+                         const float* c2, const TcBuffers& tb, int Q, int flush_tiles, int* status) {
+    const TcPlan pl = tc_plan(D, K, 148);
+    TcKernelParams p;
+    p.X = X; p.n = n; p.D = D; p.K = K; p.CL = pl.CL; p.Q = Q; p.n_ks = pl.n_ks;
+    p.flush = (flush_tiles < 2) ? 2 : (flush_tiles & ~1);
+    p.phi_img = tb.phi_img; p.plo_img = tb.plo_img; p.tk = tb.tk; p.ck = tb.ck; p.sd = tb.sd; p.kap = tb.kap;
+    p.illb = tb.illb; p.mu = mu; p.w2 = w2; p.c2 = c2;
+    p.partial = tb.partial; p.llpart = tb.llpart; p.status = status;
+#ifdef FLASHGMM_DEBUG
+    p.dbg = g_tc_debug;
+#endif
+    cudaError_t e = cudaFuncSetAttribute(em_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    if (pl.CL > 8) return cudaErrorInvalidValue;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(Q * pl.CL));
+    cfg.blockDim = dim3(NTHREADS);
+    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)pl.CL;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, em_tc_kernel, p);
+}
+
+// Number of clusters of the plan's size that can be resident at once (1 CTA per SM): the persistent grid size.
+cudaError_t tc_max_clusters(int D, int K, int* out) {
+    const TcPlan pl = tc_plan(D, K, 148);
+    cudaError_t e = cudaFuncSetAttribute(em_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(pl.CL * 148));
+    cfg.blockDim = dim3(NTHREADS);
+    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)pl.CL;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    e = cudaOccupancyMaxActiveClusters(&n, em_tc_kernel, &cfg);
+    if (e != cudaSuccess) return e;
+    *out = n;
+    return cudaSuccess;
+}
+
+cudaError_t launch_reduce_tc(cudaStream_t s, int D, int K, int Q, const TcBuffers& tb, double* Nk, double* S1,
+                             double* S2, bool accumulate) {
+    const TcPlan pl = tc_plan(D, K, 148);
+    const size_t per = (size_t)K + 2 * (size_t)K * D;
+    tc_reduce_kernel<<<(unsigned)((per + 255) / 256), 256, 0, s>>>(D, K, pl.Kpad, Q, tb.partial, tb.sd, tb.kap, Nk, S1, S2, accumulate ? 1 : 0);
+    return cudaGetLastError();
+}
+
+}  // namespace fg

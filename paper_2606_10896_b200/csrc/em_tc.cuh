@@ -1,0 +1,45 @@
+// Declarations of the tensor-core path (internal).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stddef.h>
+
+namespace fg {
+
+constexpr int TC_BN = 64;            // points per tile
+constexpr int TC_FLUSH = 64;         // tiles between flushes of the TMEM accumulators into float64 partials (even)
+constexpr float TC_RSCALE = 4096.f;  // responsibilities are scaled by this power of two before the fp16 split
+constexpr int TC_PCOLS = 257;        // columns of a partial row: 256 statistics columns + N_k
+
+struct TcPlan {
+    int CL;     // CTAs per cluster = ceil(K / 128)
+    int Kpad;   // CL * 128
+    int Q;      // clusters in the persistent grid
+    int n_ks;   // k-steps of 8 dimensions
+};
+
+struct TcBuffers {
+    uint32_t* phi_img;
+    unsigned char* plo_img;
+    float* tk;
+    float* ck;
+    float* sd;
+    float* kap;
+    float* illb;
+    double* partial;
+    double* llpart;
+};
+
+bool tc_supports(int D, int K);
+TcPlan tc_plan(int D, int K, int num_sms);
+size_t tc_scratch_bytes(int D, int K);
+cudaError_t tc_max_clusters(int D, int K, int* out);
+cudaError_t launch_prepare_tc(cudaStream_t s, int D, int K, const float* pi, const float* mu, const float* var,
+                              const TcBuffers& tb, float cond_limit, int* status);
+// mu, w2, c2: the FP32 path's derived parameters (launch_prepare_fp32), used to recompute ill-conditioned logits exactly
+cudaError_t launch_em_tc(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu, const float* w2,
+                         const float* c2, const TcBuffers& tb, int Q, int flush_tiles, int* status);
+cudaError_t launch_reduce_tc(cudaStream_t s, int D, int K, int Q, const TcBuffers& tb, double* Nk, double* S1,
+                             double* S2, bool accumulate);
+
+}  // namespace fg

@@ -1,10 +1,12 @@
 // Host side of libflashgmm: context, argument checking, scratch management, path dispatch, the EM driver and the
 // host-streaming variant.  Every step of the numerical path runs in the CUDA kernels of the other files.
 #include "internal.cuh"
+#include "em_tc.cuh"
 
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -25,7 +27,9 @@ constexpr int EVENT_POOL = 128;
 inline size_t align256(size_t b) { return (b + 255) & ~(size_t)255; }
 
 struct ScratchLayout {
-    size_t w2, c2, partials, logZ2, llpart, result, stats, derived_tc, total;
+    size_t w2, c2, partials, logZ2, llpart, result, stats, total;
+    size_t tc_phi, tc_plo, tc_tk, tc_ck, tc_sd, tc_kap, tc_illb, tc_partial, tc_llpart, tc_partial_bytes;
+    bool tc;
 };
 
 ScratchLayout scratch_layout(int D, int K) {
@@ -40,7 +44,22 @@ ScratchLayout scratch_layout(int D, int K) {
     L.llpart = take((size_t)(SUPER_TILE / FP32_TILE_P) * 8);
     L.result = take(sizeof(DevResult));
     L.stats = take(((size_t)K + 2 * KD) * 8);
-    L.derived_tc = take(0);
+    L.tc = tc_supports(D, K);
+    L.tc_phi = L.tc_plo = L.tc_tk = L.tc_ck = L.tc_sd = L.tc_kap = L.tc_illb = L.tc_partial = L.tc_llpart = 0;
+    L.tc_partial_bytes = 0;
+    if (L.tc) {
+        const TcPlan pl = tc_plan(D, K, 160);       // an upper bound on the number of clusters
+        L.tc_phi = take((size_t)pl.CL * 128 * 128 * 4);
+        L.tc_plo = take((size_t)pl.CL * 65536);
+        L.tc_tk = take((size_t)pl.Kpad * 4);
+        L.tc_ck = take((size_t)pl.Kpad * 4);
+        L.tc_sd = take(128 * 4);
+        L.tc_kap = take(128 * 4);
+        L.tc_illb = take((size_t)pl.Kpad * 4);
+        L.tc_partial_bytes = (size_t)pl.Q * pl.Kpad * TC_PCOLS * 8;
+        L.tc_partial = take(L.tc_partial_bytes);
+        L.tc_llpart = take((size_t)pl.Q * 8);
+    }
     L.total = off;
     return L;
 }
@@ -57,6 +76,9 @@ struct gmm_ctx {
     size_t scratch_bytes = 0;
     int capD = 0, capK = 0;
     ScratchLayout lay{};
+    int tc_Q = 0;              // resident clusters of the tensor-path kernel for (capD, capK)
+    float tc_cond_limit = 3e-3f;
+    int tc_flush = TC_FLUSH;
     // host-streaming path
     cudaStream_t copy_stream = nullptr;
     float* xstage[2] = {nullptr, nullptr};
@@ -80,6 +102,19 @@ struct gmm_ctx {
     double* llpart() const { return reinterpret_cast<double*>(scratch + lay.llpart); }
     DevResult* result() const { return reinterpret_cast<DevResult*>(scratch + lay.result); }
     double* stats() const { return reinterpret_cast<double*>(scratch + lay.stats); }
+    TcBuffers tc() const {
+        TcBuffers b;
+        b.phi_img = reinterpret_cast<uint32_t*>(scratch + lay.tc_phi);
+        b.plo_img = scratch + lay.tc_plo;
+        b.tk = reinterpret_cast<float*>(scratch + lay.tc_tk);
+        b.ck = reinterpret_cast<float*>(scratch + lay.tc_ck);
+        b.sd = reinterpret_cast<float*>(scratch + lay.tc_sd);
+        b.kap = reinterpret_cast<float*>(scratch + lay.tc_kap);
+        b.illb = reinterpret_cast<float*>(scratch + lay.tc_illb);
+        b.partial = reinterpret_cast<double*>(scratch + lay.tc_partial);
+        b.llpart = reinterpret_cast<double*>(scratch + lay.tc_llpart);
+        return b;
+    }
 };
 
 namespace {
@@ -131,6 +166,14 @@ int ensure_scratch(gmm_ctx* ctx, int D, int K) {
     ctx->lay = L;
     ctx->capD = D;
     ctx->capK = K;
+    ctx->tc_Q = 0;
+    if (L.tc) {
+        int q = 0;
+        CU(tc_max_clusters(D, K, &q));
+        const TcPlan pl = tc_plan(D, K, 160);
+        if (q > pl.Q) q = pl.Q;
+        ctx->tc_Q = q;
+    }
     return GMM_OK;
 }
 
@@ -183,25 +226,40 @@ int prof_end(gmm_ctx* ctx) {
     return GMM_OK;
 }
 
-int choose_path(gmm_ctx* ctx, int D, int K, int* path) {
-    (void)D; (void)K;
-    if (ctx->path == GMM_PATH_TENSOR) return fail(ctx, GMM_EUNSUPPORTED, "the tensor-core path cannot run D=%d K=%d", D, K);
-    *path = GMM_PATH_FP32;
-    return GMM_OK;
-}
-
-// Derived per-component constants for the chosen path; validates the parameters into the status word.
-int prepare_params(gmm_ctx* ctx, int path, int D, int K, const float* pi, const float* mu, const float* var) {
-    (void)path;
+// Derived per-component constants for both paths; validates the parameters into the status word.  Then picks the
+// path: the tensor-core path whenever the shape allows it (ill-conditioned components are handled inside its kernel).
+int prepare_and_choose(gmm_ctx* ctx, int D, int K, const float* pi, const float* mu, const float* var, int* path) {
     CU(cudaMemsetAsync(&ctx->result()->status, 0, sizeof(int), ctx->stream));
     KL(launch_prepare_fp32(ctx->stream, D, K, pi, mu, var, ctx->w2(), ctx->c2(), &ctx->result()->status));
+    const bool tc_ok = ctx->lay.tc && ctx->tc_Q >= 1;
+    if (ctx->path == GMM_PATH_TENSOR && !tc_ok)
+        return fail(ctx, GMM_EUNSUPPORTED, "the tensor-core path needs D <= 128 and K <= 1024 (got D=%d K=%d)", D, K);
+    if (ctx->path == GMM_PATH_FP32 || !tc_ok) {
+        *path = GMM_PATH_FP32;
+        return GMM_OK;
+    }
+    KL(launch_prepare_tc(ctx->stream, D, K, pi, mu, var, ctx->tc(), ctx->tc_cond_limit, &ctx->result()->status));
+    ctx->launches++;   // launch_prepare_tc enqueues two kernels
+    *path = GMM_PATH_TENSOR;
     return GMM_OK;
 }
 
 // Adds the statistics of n device-resident points to (Nk, S1, S2) and their log-likelihood to result()->ll[slot].
 int accumulate_points(gmm_ctx* ctx, int path, const float* X, int64_t n, int D, int K, const float* mu, double* Nk,
                       double* S1, double* S2, int slot) {
-    (void)path;
+    if (path == GMM_PATH_TENSOR) {
+        const TcBuffers tb = ctx->tc();
+        const TcPlan pl = tc_plan(D, K, 160);
+        const int Q = ctx->tc_Q;
+        CU(cudaMemsetAsync(tb.partial, 0, (size_t)Q * pl.Kpad * TC_PCOLS * 8, ctx->stream));
+        CU(cudaMemsetAsync(tb.llpart, 0, (size_t)Q * 8, ctx->stream));
+        CHECK(prof_begin(ctx));
+        KL(launch_em_tc(ctx->stream, X, n, D, K, mu, ctx->w2(), ctx->c2(), tb, Q, ctx->tc_flush, &ctx->result()->status));
+        CHECK(prof_end(ctx));
+        KL(launch_reduce_ll(ctx->stream, tb.llpart, Q, &ctx->result()->ll[slot], true));
+        KL(launch_reduce_tc(ctx->stream, D, K, Q, tb, Nk, S1, S2, true));
+        return GMM_OK;
+    }
     const Fp32Plan plan = fp32_plan(D, K);
     for (int64_t off = 0; off < n; off += SUPER_TILE) {
         const int64_t cnt = (n - off < SUPER_TILE) ? (n - off) : SUPER_TILE;
@@ -267,6 +325,8 @@ int gmm_create(gmm_ctx** out, int device, void* cuda_stream) {
     if (!ctx) return GMM_ENOMEM;
     ctx->device = device;
     ctx->stream = static_cast<cudaStream_t>(cuda_stream);
+    if (const char* e = std::getenv("GMM_TC_COND_LIMIT")) ctx->tc_cond_limit = (float)std::atof(e);
+    if (const char* e = std::getenv("GMM_TC_FLUSH")) ctx->tc_flush = std::atoi(e);
     *out = ctx;
     return GMM_OK;
 }
@@ -316,9 +376,8 @@ int gmm_em_step(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const flo
     if (!loglik) return fail(ctx, GMM_EINVAL, "loglik is NULL");
     DeviceGuard g(ctx->device);
     int path;
-    CHECK(choose_path(ctx, D, K, &path));
     CHECK(ensure_scratch(ctx, D, K));
-    CHECK(prepare_params(ctx, path, D, K, pi, mu, var));
+    CHECK(prepare_and_choose(ctx, D, K, pi, mu, var, &path));
     CHECK(zero_stats(ctx, D, K, Nk, S1, S2, 0));
     CHECK(accumulate_points(ctx, path, X, N, D, K, mu, Nk, S1, S2, 0));
     ctx->last_path = path;
@@ -353,7 +412,6 @@ int gmm_fit(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, float* pi, fl
     if (!(tol >= 0.0)) return fail(ctx, GMM_EINVAL, "tol must be >= 0");
     DeviceGuard g(ctx->device);
     int path;
-    CHECK(choose_path(ctx, D, K, &path));
     CHECK(ensure_scratch(ctx, D, K));
     const size_t KD = (size_t)K * D;
     double* Nk = ctx->stats();
@@ -362,7 +420,7 @@ int gmm_fit(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, float* pi, fl
     int t = 0;
     for (; t < iters; ++t) {
         const int slot = t % LL_SLOTS;
-        CHECK(prepare_params(ctx, path, D, K, pi, mu, var));
+        CHECK(prepare_and_choose(ctx, D, K, pi, mu, var, &path));
         CHECK(zero_stats(ctx, D, K, Nk, S1, S2, slot));
         CHECK(accumulate_points(ctx, path, X, N, D, K, mu, Nk, S1, S2, slot));
         KL(launch_finalize(ctx->stream, N, D, K, Nk, S1, S2, var_floor, pi, mu, var));
@@ -396,7 +454,6 @@ int gmm_em_step_host(gmm_ctx* ctx, const float* X_host, int64_t N, int D, int K,
     if (!loglik) return fail(ctx, GMM_EINVAL, "loglik is NULL");
     DeviceGuard g(ctx->device);
     int path;
-    CHECK(choose_path(ctx, D, K, &path));
     CHECK(ensure_scratch(ctx, D, K));
     const size_t KD = (size_t)K * D;
     // one-time resources of the host path
@@ -437,7 +494,7 @@ int gmm_em_step_host(gmm_ctx* ctx, const float* X_host, int64_t N, int D, int K,
     double* Nk = ctx->stats();
     double* S1 = Nk + K;
     double* S2 = S1 + KD;
-    CHECK(prepare_params(ctx, path, D, K, pi, mu, var));
+    CHECK(prepare_and_choose(ctx, D, K, pi, mu, var, &path));
     CHECK(zero_stats(ctx, D, K, Nk, S1, S2, 0));
     const int64_t rows_per_chunk = (int64_t)(STAGE_BYTES / ((size_t)D * 4));
     if (rows_per_chunk < 1) return fail(ctx, GMM_EINVAL, "D too large for the staging buffer");
@@ -471,7 +528,8 @@ int gmm_assign_topm(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const
     if (m < 1 || m > K || m > GMM_MAX_TOPM) return fail(ctx, GMM_EINVAL, "m must be in [1, min(K, %d)] (got %d)", GMM_MAX_TOPM, m);
     DeviceGuard g(ctx->device);
     CHECK(ensure_scratch(ctx, D, K));
-    CHECK(prepare_params(ctx, GMM_PATH_FP32, D, K, pi, mu, var));
+    CU(cudaMemsetAsync(&ctx->result()->status, 0, sizeof(int), ctx->stream));
+    KL(launch_prepare_fp32(ctx->stream, D, K, pi, mu, var, ctx->w2(), ctx->c2(), &ctx->result()->status));
     for (int64_t off = 0; off < N; off += SUPER_TILE) {
         const int64_t cnt = (N - off < SUPER_TILE) ? (N - off) : SUPER_TILE;
         KL(launch_topm_fp32(ctx->stream, X + off * D, cnt, D, K, mu, ctx->w2(), ctx->c2(), m, idx + off * m, resp + off * m));
@@ -479,6 +537,8 @@ int gmm_assign_topm(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const
     ctx->last_path = GMM_PATH_FP32;
     return GMM_OK;
 }
+
+int gmm_tensor_path_supports(int D, int K) { return tc_supports(D, K) ? 1 : 0; }
 
 size_t gmm_scratch_bytes(int D, int K) {
     if (D < 1 || K < 1) return 0;

@@ -17,7 +17,7 @@ constexpr int FP32_TARGET_CTAS = 296;
 constexpr int LL_SLOTS = 64;       // device slots for log-likelihood values (gmm_fit keeps one per iteration in a ring)
 
 // Status word bits written by device code, read by the host after a synchronising call.
-enum : int { ST_BAD_VAR = 1, ST_BAD_PI = 2, ST_NONFINITE = 4, ST_TIMEOUT = 8 };
+enum : int { ST_BAD_VAR = 1, ST_BAD_PI = 2, ST_NONFINITE = 4, ST_TIMEOUT = 8, ST_ILLCOND = 16 };
 
 struct Fp32Plan {
     int comp_blocks, d_chunks, splits;

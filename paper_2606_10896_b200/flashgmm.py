@@ -26,6 +26,7 @@ EXPORTS = {
     "gmm_destroy": (ctypes.c_int, [ctypes.c_void_p]),
     "gmm_set_path": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int]),
     "gmm_last_path": (ctypes.c_int, [ctypes.c_void_p]),
+    "gmm_tensor_path_supports": (ctypes.c_int, [ctypes.c_int, ctypes.c_int]),
     "gmm_em_step": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_int,
                                    ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                    ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
@@ -80,6 +81,10 @@ class GmmError(RuntimeError):
     def __init__(self, code: int, message: str):
         super().__init__(f"libflashgmm error {code} ({lib.gmm_strerror(code).decode()}): {message}")
         self.code = code
+
+
+def tensor_path_supports(D: int, K: int) -> bool:
+    return bool(lib.gmm_tensor_path_supports(int(D), int(K)))
 
 
 def gmm_scratch_bytes(D: int, K: int) -> int:

@@ -33,9 +33,11 @@ namespace fg {
 namespace {
 
 constexpr int BN = TC_BN;                 // points per tile
-constexpr int NTHREADS = 288;
+constexpr int NTHREADS = 416;          // 2 softmax warpgroups (even / odd tiles), 1 transform warpgroup, 1 MMA warp
+constexpr int MMA_WARP = 12;
 constexpr float RSCALE = TC_RSCALE;
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
+constexpr float ILL_ABS = 1000.f;
 
 // shared memory map (offsets from a 1024-byte aligned base)
 constexpr int SM_PLO = 0;                       // 65536
@@ -43,19 +45,27 @@ constexpr int SM_Y = 65536;                     // 2 stages x (hi 32768 + lo 327
 constexpr int SM_YSTAGE = 65536;
 constexpr int SM_YLO = 32768;
 constexpr int SM_MISC = SM_Y + 2 * SM_YSTAGE;   // 196608
-constexpr int SM_GATHER = SM_MISC;              // 4 warps x 64 floats           1024
-constexpr int SM_WS = SM_GATHER + 1024;         // 4 warps x 64 float2           2048
-constexpr int SM_FAC = SM_WS + 2048;            // 4 warps x 64 floats           1024
-constexpr int SM_EXCH = SM_FAC + 1024;          // 2 bufs x 8 CTAs x 64 float2   8192
+constexpr int SM_GATHER = SM_MISC;              // 2 groups x 4 warps x 64 floats    2048
+constexpr int SM_WS = SM_GATHER + 2048;         // 2 groups x 4 warps x 64 float2    4096
+constexpr int SM_FAC = SM_WS + 4096;            // 2 groups x 4 warps x 64 floats    2048
+constexpr int SM_EXCH = SM_FAC + 2048;          // 2 bufs x 8 CTAs x 64 float2       8192
 constexpr int SM_SD = SM_EXCH + 8192;           // 128 floats                     512
 constexpr int SM_KAP = SM_SD + 512;             // 128 floats                     512
-constexpr int SM_LL = SM_KAP + 512;             // 64 doubles                     512
-constexpr int SM_BAR = SM_LL + 512;             // barriers                       256
+constexpr int SM_LL = SM_KAP + 512;             // 2 x 64 doubles                1024
+constexpr int SM_BAR = SM_LL + 1024;             // barriers                       256
 constexpr int SM_END = SM_BAR + 256;
 constexpr int SMEM_BYTES = SM_END + 1024;       // + alignment slack
 
 enum { B_YFULL0 = 0, B_YFULL1, B_YEMPTY0, B_YEMPTY1, B_LFULL0, B_LFULL1, B_RREADY0, B_RREADY1, B_X0, B_X1, B_ACCFULL,
        B_ACCFREE, B_FINAL, B_COUNT };
+
+#ifdef FLASHGMM_DEBUG
+#define TIC(var) long long var = clock64()
+#define TOC(var, slot) do { if (p.dbg_clk && blockIdx.x == 0) { long long now_ = clock64(); if ((threadIdx.x & 31) == 0) atomicAdd((unsigned long long*)&p.dbg_clk[slot], (unsigned long long)(now_ - var)); var = now_; } } while (0)
+#else
+#define TIC(var)
+#define TOC(var, slot)
+#endif
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -123,6 +133,14 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t cta
 }
 __device__ __forceinline__ void st_remote_f2(uint32_t remote_addr, float a, float b) {
     asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(remote_addr), "f"(a), "f"(b) : "memory");
+}
+// Remote 8-byte store that signals the destination CTA's mbarrier with its byte count (no release round trip).
+__device__ __forceinline__ void st_async_f2(uint32_t remote_addr, float a, float b, uint32_t remote_bar) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.f32 [%0], {%1, %2}, [%3];"
+                 ::"r"(remote_addr), "f"(a), "f"(b), "r"(remote_bar) : "memory");
+}
+__device__ __forceinline__ void bar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ uint32_t cluster_rank() {
     uint32_t r;
@@ -230,7 +248,8 @@ struct TcKernelParams {
     double* llpart;                // [Q]
     int* status;
 #ifdef FLASHGMM_DEBUG
-    float* dbg;      // [Kpad][64] log2 z of the first tile, [Kpad][64] r of the first tile
+    float* dbg;      // [Kpad][64] log2 z of the first tile
+    long long* dbg_clk;   // per-phase cycle counters of CTA 0
 #endif
 };
 
@@ -239,7 +258,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
     unsigned char* smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
-    __shared__ int decision_s;
+    __shared__ int decision_s[2];
     volatile int* abort_flag = &abort_s;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -255,17 +274,18 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
 
     if (tid == 0) {
         abort_s = 0;
-        decision_s = 0;
+        decision_s[0] = 0;
+        decision_s[1] = 0;
         bar_init(BAR(B_YFULL0), 128);  bar_init(BAR(B_YFULL1), 128);
         bar_init(BAR(B_YEMPTY0), 1);   bar_init(BAR(B_YEMPTY1), 1);
         bar_init(BAR(B_LFULL0), 1);    bar_init(BAR(B_LFULL1), 1);
         bar_init(BAR(B_RREADY0), 128); bar_init(BAR(B_RREADY1), 128);
-        bar_init(BAR(B_X0), p.CL * 64); bar_init(BAR(B_X1), p.CL * 64);
+        bar_init(BAR(B_X0), 1); bar_init(BAR(B_X1), 1);
         bar_init(BAR(B_ACCFULL), 1);   bar_init(BAR(B_ACCFREE), 128);
         bar_init(BAR(B_FINAL), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 8) {
+    if (warp == MMA_WARP) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(512) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -304,33 +324,37 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
     fence_after();
     if (p.CL > 1) cluster_sync_all();      // peers' barriers are initialised before anyone sends to them
 
-    if (warp < 4) {
+    if (warp < 8) {
         // =========================== softmax warps ===========================
-        const uint32_t lane_addr = ((uint32_t)(warp * 32)) << 16;
-        const int kloc = tid;                                   // component within the slice
+        // Two warpgroups: group g (warps 4g..4g+3) handles the local tiles with i % 2 == g, i.e. always stage / logits
+        // buffer g, so a tile's softmax has two tile periods of the tensor pipe to finish.
+        const int grp = warp >> 2, wq = warp & 3, gtid = tid & 127;
+        const uint32_t lane_addr = ((uint32_t)(wq * 32)) << 16;
+        const int kloc = gtid;                                  // component within the slice
         const float tk = p.tk[rank * 128 + kloc];
         const float ck = p.ck[rank * 128 + kloc];
         const float illb = p.illb[rank * 128 + kloc];
         float* gather = reinterpret_cast<float*>(smem + SM_GATHER) + warp * 64;
-        float2* ws = reinterpret_cast<float2*>(smem + SM_WS);          // [4][64]
-        float* fac = reinterpret_cast<float*>(smem + SM_FAC);          // [4][64]
+        float2* ws = reinterpret_cast<float2*>(smem + SM_WS) + grp * 256;      // [4][64] per group
+        float* fac = reinterpret_cast<float*>(smem + SM_FAC) + grp * 256;      // [4][64] per group
         float2* exch = reinterpret_cast<float2*>(smem + SM_EXCH);      // [2][8][64]
         float nk_acc = 0.f;
         double ll_acc = 0.0;
         double* prow = p.partial + ((size_t)cluster_id * (p.CL * 128) + rank * 128 + kloc) * TC_PCOLS;
-        uint32_t accfull_parity = 0;
         bool alive = true;
 
         // Softmax threads leave the loop only at the uniform decision point after named barrier 2: a thread that
         // left earlier would strand the others in a hardware barrier.
-        for (int64_t i = 0; i < ntl; ++i) {
-            const int s = (int)(i & 1);
+        for (int64_t i = grp; i < ntl; i += 2) {
+            const int s = grp;
             const uint32_t ph = (uint32_t)((i >> 1) & 1);
             const int64_t tile = cluster_id + i * p.Q;
             const int64_t row0 = tile * BN;
             const int nvalid = (int)((p.n - row0 < BN) ? (p.n - row0) : BN);
 
+            TIC(tk_);
             if (!bar_wait(BAR(B_LFULL0 + s), ph, abort_flag, p.status, false)) alive = false;
+            TOC(tk_, 0);
             fence_after();
             float l[64];
             {
@@ -348,6 +372,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
             if (p.dbg && cluster_id == 0 && i == 0)
                 for (int j = 0; j < 64; ++j) p.dbg[(size_t)(rank * 128 + kloc) * 64 + j] = l[j];
 #endif
+            TOC(tk_, 16);
             // warp-level max per point, all-gathered through shared memory
             float red[2];
             warp_reduce_scatter<true>(l, red, lane);
@@ -360,10 +385,15 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
             if (__any_sync(0xffffffffu, illb > 0.f)) {
                 uint32_t mlo = 0, mhi = 0;
                 if (illb > 0.f) {
+                    // Two conditions: within `illb` of the warp's best logit for the point, and not absurdly far from the
+                    // component in absolute terms (log2 z - c_k = -log2e/2 * Mahalanobis^2 >= -ILL_ABS, about ten times the
+                    // expected D/2): the second one keeps ordinary points of other components, for which every
+                    // component of this warp is equally hopeless, out of the exact path.
+                    const float floor_abs = ck - ILL_ABS - illb;
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
-                        if (j < nvalid && l[j] >= gather[j] - illb) mlo |= 1u << j;
-                        if (32 + j < nvalid && l[32 + j] >= gather[32 + j] - illb) mhi |= 1u << j;
+                        if (l[j] >= floor_abs && j < nvalid && l[j] >= gather[j] - illb) mlo |= 1u << j;
+                        if (l[32 + j] >= floor_abs && 32 + j < nvalid && l[32 + j] >= gather[32 + j] - illb) mhi |= 1u << j;
                     }
                 }
                 bool fixed_any = false;
@@ -401,6 +431,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                     __syncwarp();
                 }
             }
+            TOC(tk_, 17);
             const float mw_mine0 = red[0], mw_mine1 = red[1];
 #pragma unroll
             for (int j = 0; j < 64; j += 4) {
@@ -415,12 +446,15 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                 l[j + 3] = fast_ex2(l[j + 3] - m3);
             }
             __syncwarp();
+            TOC(tk_, 18);
             float sred[2];
             warp_reduce_scatter<false>(l, sred, lane);
-            *reinterpret_cast<float4*>(&ws[warp * 64 + 2 * lane]) = make_float4(mw_mine0, sred[0], mw_mine1, sred[1]);
-            named_bar_sync(1, 128);
-            if (tid < 64) {
-                const int pt = tid;
+            *reinterpret_cast<float4*>(&ws[wq * 64 + 2 * lane]) = make_float4(mw_mine0, sred[0], mw_mine1, sred[1]);
+            TOC(tk_, 1);
+            named_bar_sync(1 + 2 * grp, 128);
+            TOC(tk_, 2);
+            if (gtid < 64) {
+                const int pt = gtid;
                 float2 w4[4];
 #pragma unroll
                 for (int w = 0; w < 4; ++w) w4[w] = ws[w * 64 + pt];
@@ -432,11 +466,11 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                     sc += (w4[w].x == -CUDART_INF_F) ? 0.f : w4[w].y * fast_ex2(w4[w].x - mc_safe);
                 // send (m, s) of this CTA's 128 components to every CTA of the cluster (including this one)
                 const uint32_t slot = smem_u32(&exch[(s * 8 + rank) * 64 + pt]);
-                for (int c = 0; c < p.CL; ++c) {
-                    st_remote_f2(map_to_cta(slot, c), mc, sc);
-                    bar_arrive_remote(map_to_cta(BAR(B_X0 + s), c));
-                }
-                if (!bar_wait(BAR(B_X0 + s), ph, abort_flag, p.status, true)) alive = false;
+                if (pt == 0) bar_arrive_expect_tx(BAR(B_X0 + s), (uint32_t)p.CL * 64u * 8u);   // this tile's incoming bytes
+                for (int c = 0; c < p.CL; ++c) st_async_f2(map_to_cta(slot, c), mc, sc, map_to_cta(BAR(B_X0 + s), c));
+                TOC(tk_, 3);
+                if (!bar_wait(BAR(B_X0 + s), ph, abort_flag, p.status, false)) alive = false;
+                TOC(tk_, 4);
                 float mi = -CUDART_INF_F;
                 float2 e[8];
 #pragma unroll
@@ -456,26 +490,29 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                     fac[w * 64 + pt] = (w4[w].x == -CUDART_INF_F) ? 0.f : fast_ex2(w4[w].x - mi_safe) * inv;
                 if (rank == 0 && valid) ll_acc += (double)(mi + log2f(Z));
             }
-            if (tid == 0) decision_s = *abort_flag;
-            named_bar_sync(2, 128);
-            if (decision_s) break;
+            if (gtid == 0) decision_s[grp] = *abort_flag;
+            TOC(tk_, 5);
+            named_bar_sync(2 + 2 * grp, 128);
+            TOC(tk_, 6);
+            if (decision_s[grp]) break;
             // responsibilities: r = p * fac, split into fp16 hi + lo, written over the logits as the M-step A operand
             {
                 uint32_t hi[32], lo[32];
-                const float* fw = fac + warp * 64;
+                const float* fw = fac + wq * 64;
                 float nsum = 0.f;
 #pragma unroll
                 for (int j = 0; j < 64; j += 4) {
                     const float4 f4 = *reinterpret_cast<const float4*>(fw + j);
                     const float r0 = l[j] * f4.x, r1 = l[j + 1] * f4.y, r2 = l[j + 2] * f4.z, r3 = l[j + 3] * f4.w;
-                    const __half h0 = __float2half_rn(r0), h1 = __float2half_rn(r1), h2 = __float2half_rn(r2), h3 = __float2half_rn(r3);
-                    const float b0 = __half2float(h0), b1 = __half2float(h1), b2 = __half2float(h2), b3 = __half2float(h3);
-                    const __half g0 = __float2half_rn(r0 - b0), g1 = __float2half_rn(r1 - b1), g2 = __float2half_rn(r2 - b2), g3 = __float2half_rn(r3 - b3);
-                    nsum += (b0 + __half2float(g0)) + (b1 + __half2float(g1)) + (b2 + __half2float(g2)) + (b3 + __half2float(g3));
-                    hi[j / 2] = pack_h2(h0, h1);
-                    hi[j / 2 + 1] = pack_h2(h2, h3);
-                    lo[j / 2] = pack_h2(g0, g1);
-                    lo[j / 2 + 1] = pack_h2(g2, g3);
+                    const __half2 h01 = __floats2half2_rn(r0, r1), h23 = __floats2half2_rn(r2, r3);
+                    const float2 b01 = __half22float2(h01), b23 = __half22float2(h23);
+                    const __half2 g01 = __floats2half2_rn(r0 - b01.x, r1 - b01.y), g23 = __floats2half2_rn(r2 - b23.x, r3 - b23.y);
+                    const float2 c01 = __half22float2(g01), c23 = __half22float2(g23);
+                    nsum += ((b01.x + c01.x) + (b01.y + c01.y)) + ((b23.x + c23.x) + (b23.y + c23.y));
+                    hi[j / 2] = *reinterpret_cast<const uint32_t*>(&h01);
+                    hi[j / 2 + 1] = *reinterpret_cast<const uint32_t*>(&h23);
+                    lo[j / 2] = *reinterpret_cast<const uint32_t*>(&g01);
+                    lo[j / 2 + 1] = *reinterpret_cast<const uint32_t*>(&g23);
                 }
                 nk_acc += nsum;
                 tmem_st32(T_LOG + s * 64 + lane_addr, hi);
@@ -484,13 +521,15 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
             }
             fence_before();
             bar_arrive(BAR(B_RREADY0 + s));
+            TOC(tk_, 7);
 
-            // periodic flush of the TMEM accumulators into float64 partials (after the second tile of a pair)
+            // periodic flush of the TMEM accumulators into float64 partials: by the group that owns the last tile of the
+            // pair; the flush index (hence the barrier parity) follows from the tile index alone
             const bool pair_end = (i & 1) || (i + 1 == ntl);
             const int64_t pair_next = (i | 1) + 1;
             if (pair_end && ((pair_next % p.flush) == 0 || pair_next >= ntl)) {
-                if (!bar_wait(BAR(B_ACCFULL), accfull_parity, abort_flag, p.status, false)) alive = false;
-                accfull_parity ^= 1;
+                const uint32_t fpar = (uint32_t)(((pair_next - 1) / p.flush) & 1);
+                if (!bar_wait(BAR(B_ACCFULL), fpar, abort_flag, p.status, false)) alive = false;
                 fence_after();
 #pragma unroll 1
                 for (int c0 = 0; c0 < 256; c0 += 32) {
@@ -500,25 +539,29 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
 #pragma unroll
                     for (int j = 0; j < 32; ++j) prow[c0 + j] += (double)__uint_as_float(v[j]);
                 }
-                prow[256] += (double)nk_acc;
-                nk_acc = 0.f;
                 fence_before();
                 bar_arrive(BAR(B_ACCFREE));
+                TOC(tk_, 8);
+            }
+            // N_k of this group's tiles has its own column, flushed on the group's own cadence
+            if ((((i >> 1) + 1) % 32) == 0 || i + 2 >= ntl) {
+                prow[256 + grp] += (double)nk_acc;
+                nk_acc = 0.f;
             }
         }
         if (rank == 0) {
-            double* lls = reinterpret_cast<double*>(smem + SM_LL);
-            if (tid < 64) lls[tid] = ll_acc;
-            named_bar_sync(3, 128);
-            if (tid == 0) {
+            double* lls = reinterpret_cast<double*>(smem + SM_LL) + grp * 64;
+            if (gtid < 64) lls[gtid] = ll_acc;
+            named_bar_sync(5 + grp, 128);
+            if (gtid == 0) {
                 double sum = 0.0;
                 for (int j = 0; j < 64; ++j) sum += lls[j];
-                p.llpart[cluster_id] = sum * 0.69314718055994530942;
+                p.llpart[cluster_id * 2 + grp] = sum * 0.69314718055994530942;
             }
         }
-    } else if (warp < 8) {
+    } else if (warp < MMA_WARP) {
         // =========================== transform warps: X -> Y planes ===========================
-        const int tau = tid - 128;
+        const int tau = tid - 256;
         const int pt = tau >> 1, half = tau & 1;
         const bool vec_ok = (p.D % 4 == 0) && ((reinterpret_cast<uintptr_t>(p.X) & 15) == 0);
         for (int64_t i = 0; i < ntl; ++i) {
@@ -527,24 +570,38 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
             const int64_t row = (cluster_id + i * p.Q) * BN + pt;
             const bool row_ok = row < p.n;
             const float* xr = p.X + row * p.D;
+            unsigned char* yhi = smem + SM_Y + s * SM_YSTAGE;
+            unsigned char* ylo = yhi + SM_YLO;
+            float4 xa[8], xb[8];
+            const bool fast = row_ok && vec_ok && (half * 64 + 64 <= p.D);
+            if (fast) {
+#pragma unroll
+                for (int g = 0; g < 8; ++g) {
+                    xa[g] = __ldg(reinterpret_cast<const float4*>(xr + half * 64 + g * 8));
+                    xb[g] = __ldg(reinterpret_cast<const float4*>(xr + half * 64 + g * 8 + 4));
+                }
+            } else {
+#pragma unroll
+                for (int g = 0; g < 8; ++g) {
+                    const int d0 = half * 64 + g * 8;
+                    float x[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) x[j] = (row_ok && d0 + j < p.D) ? __ldg(xr + d0 + j) : 0.f;
+                    xa[g] = make_float4(x[0], x[1], x[2], x[3]);
+                    xb[g] = make_float4(x[4], x[5], x[6], x[7]);
+                }
+            }
+            // the loads above are in flight while this thread waits for the stage to be released
+            TIC(tt_);
             if (i >= 2) {
                 if (!bar_wait(BAR(B_YEMPTY0 + s), ph ^ 1, abort_flag, p.status, false)) break;
             }
-            unsigned char* yhi = smem + SM_Y + s * SM_YSTAGE;
-            unsigned char* ylo = yhi + SM_YLO;
-#pragma unroll 2
+            TOC(tt_, 10);
+#pragma unroll
             for (int g = 0; g < 8; ++g) {
                 const int ks = half * 8 + g;
                 const int d0 = ks * 8;
-                float x[8];
-                if (row_ok && vec_ok && d0 + 8 <= p.D) {
-                    const float4 a = __ldg(reinterpret_cast<const float4*>(xr + d0));
-                    const float4 b = __ldg(reinterpret_cast<const float4*>(xr + d0 + 4));
-                    x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
-                } else {
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) x[j] = (row_ok && d0 + j < p.D) ? __ldg(xr + d0 + j) : 0.f;
-                }
+                const float x[8] = {xa[g].x, xa[g].y, xa[g].z, xa[g].w, xb[g].x, xb[g].y, xb[g].z, xb[g].w};
                 uint32_t xh[4], xl[4], qh[4], ql[4];
 #pragma unroll
                 for (int j = 0; j < 8; j += 2) {
@@ -552,14 +609,16 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                     u0 = fminf(fmaxf(u0, -240.f), 240.f);
                     u1 = fminf(fmaxf(u1, -240.f), 240.f);
                     const float q0 = fmaf(u0, u0, kap_s[d0 + j]), q1 = fmaf(u1, u1, kap_s[d0 + j + 1]);
-                    const __half h0 = __float2half_rn(u0), h1 = __float2half_rn(u1);
-                    const __half g0 = __float2half_rn(u0 - __half2float(h0)), g1 = __float2half_rn(u1 - __half2float(h1));
-                    const __half s0 = __float2half_rn(q0), s1 = __float2half_rn(q1);
-                    const __half t0 = __float2half_rn(q0 - __half2float(s0)), t1 = __float2half_rn(q1 - __half2float(s1));
-                    xh[j / 2] = pack_h2(h0, h1);
-                    xl[j / 2] = pack_h2(g0, g1);
-                    qh[j / 2] = pack_h2(s0, s1);
-                    ql[j / 2] = pack_h2(t0, t1);
+                    const __half2 h = __floats2half2_rn(u0, u1);
+                    const float2 hf = __half22float2(h);
+                    const __half2 g2 = __floats2half2_rn(u0 - hf.x, u1 - hf.y);
+                    const __half2 sq = __floats2half2_rn(q0, q1);
+                    const float2 sf = __half22float2(sq);
+                    const __half2 t2 = __floats2half2_rn(q0 - sf.x, q1 - sf.y);
+                    xh[j / 2] = *reinterpret_cast<const uint32_t*>(&h);
+                    xl[j / 2] = *reinterpret_cast<const uint32_t*>(&g2);
+                    qh[j / 2] = *reinterpret_cast<const uint32_t*>(&sq);
+                    ql[j / 2] = *reinterpret_cast<const uint32_t*>(&t2);
                 }
                 // 16-byte chunk index in the point's 512-byte row: 2 ks (x) and 2 ks + 1 (x^2)
                 const int atom = ks >> 2;
@@ -573,6 +632,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
             }
             fence_async_smem();
             bar_arrive(BAR(B_YFULL0 + s));
+            TOC(tt_, 11);
         }
     } else if (lane == 0) {
         // =========================== MMA issuer (one thread) ===========================
@@ -585,24 +645,31 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
         auto issue_E = [&](int64_t i) -> bool {
             const int s = (int)(i & 1);
             const uint32_t ph = (uint32_t)((i >> 1) & 1);
+            TIC(tm_);
             if (!bar_wait(BAR(B_YFULL0 + s), ph, abort_flag, p.status, false)) return false;
+            TOC(tm_, 12);
             fence_after();
             const uint32_t yhi = smem_u32(smem + SM_Y + s * SM_YSTAGE), ylo = yhi + SM_YLO;
             const uint32_t d = T_LOG + s * 64;
+            // The two small cross products go first: the accumulator truncates (toward zero) at every add, by up to one
+            // ulp of its CURRENT magnitude, so they are added while it is still small.
             for (int ks = 0; ks < p.n_ks; ++ks)
-                mma_ts(d, T_PHI + ks * 8, make_desc(yhi + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024), id_e, ks > 0);
+                mma_ss(d, make_desc(plo + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024),
+                       make_desc(yhi + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024), id_e, ks > 0);
             for (int ks = 0; ks < p.n_ks; ++ks)
                 mma_ts(d, T_PHI + ks * 8, make_desc(ylo + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024), id_e, 1);
             for (int ks = 0; ks < p.n_ks; ++ks)
-                mma_ss(d, make_desc(plo + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024),
-                       make_desc(yhi + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024), id_e, 1);
+                mma_ts(d, T_PHI + ks * 8, make_desc(yhi + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024), id_e, 1);
             mma_commit(BAR(B_LFULL0 + s));
+            TOC(tm_, 13);
             return true;
         };
         auto issue_M = [&](int64_t i) -> bool {
             const int s = (int)(i & 1);
             const uint32_t ph = (uint32_t)((i >> 1) & 1);
+            TIC(tm_);
             if (!bar_wait(BAR(B_RREADY0 + s), ph, abort_flag, p.status, false)) return false;
+            TOC(tm_, 14);
             fence_after();
             const uint32_t yhi = smem_u32(smem + SM_Y + s * SM_YSTAGE), ylo = yhi + SM_YLO;
             const uint32_t rhi = T_LOG + s * 64, rlo = rhi + 32;
@@ -613,6 +680,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
             for (int ks = 0; ks < BN / 16; ++ks) mma_ts(T_ACC, rhi + ks * 8, make_desc(ylo + ks * 2048, 8192, 1024), id_m, 1);
             for (int ks = 0; ks < BN / 16; ++ks) mma_ts(T_ACC, rlo + ks * 8, make_desc(yhi + ks * 2048, 8192, 1024), id_m, 1);
             mma_commit(BAR(B_YEMPTY0 + s));
+            TOC(tm_, 15);
             return true;
         };
         for (int64_t i = 0; i < ntl && alive; i += 2) {
@@ -640,7 +708,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
     fence_before();
     __syncthreads();
     if (p.CL > 1) cluster_sync_all();
-    if (warp == 8) {
+    if (warp == MMA_WARP) {
         fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512) : "memory");
     }
@@ -769,7 +837,7 @@ __global__ void tc_reduce_kernel(int D, int K, int Kpad, int Q, const double* __
     double unscale = 1.0 / (double)TC_RSCALE;
     double* dst;
     if (e < (size_t)K) {
-        k = (int)e; col = 256; dst = Nk + e;
+        k = (int)e; col = 256; dst = Nk + e;     // plus column 257 (second softmax group), added below
     } else if (e < K + KD) {
         const size_t j = e - K; k = (int)(j / D); const int d = (int)(j % D);
         col = 16 * (d >> 3) + (d & 7); unscale /= (double)sd[d]; dst = S1 + j;
@@ -779,10 +847,12 @@ __global__ void tc_reduce_kernel(int D, int K, int Kpad, int Q, const double* __
     }
     double s = 0.0;
     for (int q = 0; q < Q; ++q) s += partial[((size_t)q * Kpad + k) * TC_PCOLS + col];
+    if (e < (size_t)K)
+        for (int q = 0; q < Q; ++q) s += partial[((size_t)q * Kpad + k) * TC_PCOLS + 257];
     if (e >= K + KD) {          // squares were accumulated as (s x)^2 + kap: take kap * N_k out again
         const int d = (int)((e - K - KD) % D);
         double nk = 0.0;
-        for (int q = 0; q < Q; ++q) nk += partial[((size_t)q * Kpad + k) * TC_PCOLS + 256];
+        for (int q = 0; q < Q; ++q) nk += partial[((size_t)q * Kpad + k) * TC_PCOLS + 256] + partial[((size_t)q * Kpad + k) * TC_PCOLS + 257];
         s -= (double)kap[d] * nk;
     }
     s *= unscale;
@@ -793,7 +863,9 @@ __global__ void tc_reduce_kernel(int D, int K, int Kpad, int Q, const double* __
 
 #ifdef FLASHGMM_DEBUG
 float* g_tc_debug = nullptr;
+long long* g_tc_clk = nullptr;
 extern "C" void gmm_debug_set_buffer(float* p) { g_tc_debug = p; }
+extern "C" void gmm_debug_set_clk(long long* p) { g_tc_clk = p; }
 #endif
 
 bool tc_supports(int D, int K) { return D >= 1 && D <= 128 && K >= 1 && K <= 1024; }
@@ -816,7 +888,7 @@ size_t tc_scratch_bytes(int D, int K) {
     b += (size_t)pl.CL * 65536;                            // P_lo image
     b += (size_t)pl.Kpad * 4 * 2 + 512;                    // t_k, c_k, s_d
     b += (size_t)pl.Q * pl.Kpad * TC_PCOLS * 8;            // float64 partials
-    b += (size_t)pl.Q * 8;
+    b += (size_t)pl.Q * 16;
     return b + 8 * 256;
 }
 
@@ -841,6 +913,7 @@ cudaError_t launch_em_tc(cudaStream_t s, const float* X, int64_t n, int D, int K
     p.partial = tb.partial; p.llpart = tb.llpart; p.status = status;
 #ifdef FLASHGMM_DEBUG
     p.dbg = g_tc_debug;
+    p.dbg_clk = g_tc_clk;
 #endif
     cudaError_t e = cudaFuncSetAttribute(em_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e != cudaSuccess) return e;

@@ -9,7 +9,7 @@ namespace fg {
 constexpr int TC_BN = 64;            // points per tile
 constexpr int TC_FLUSH = 64;         // tiles between flushes of the TMEM accumulators into float64 partials (even)
 constexpr float TC_RSCALE = 4096.f;  // responsibilities are scaled by this power of two before the fp16 split
-constexpr int TC_PCOLS = 257;        // columns of a partial row: 256 statistics columns + N_k
+constexpr int TC_PCOLS = 258;        // columns of a partial row: 256 statistics columns + N_k of each softmax group
 
 struct TcPlan {
     int CL;     // CTAs per cluster = ceil(K / 128)

@@ -58,7 +58,7 @@ ScratchLayout scratch_layout(int D, int K) {
         L.tc_illb = take((size_t)pl.Kpad * 4);
         L.tc_partial_bytes = (size_t)pl.Q * pl.Kpad * TC_PCOLS * 8;
         L.tc_partial = take(L.tc_partial_bytes);
-        L.tc_llpart = take((size_t)pl.Q * 8);
+        L.tc_llpart = take((size_t)pl.Q * 16);
     }
     L.total = off;
     return L;
@@ -252,11 +252,11 @@ int accumulate_points(gmm_ctx* ctx, int path, const float* X, int64_t n, int D, 
         const TcPlan pl = tc_plan(D, K, 160);
         const int Q = ctx->tc_Q;
         CU(cudaMemsetAsync(tb.partial, 0, (size_t)Q * pl.Kpad * TC_PCOLS * 8, ctx->stream));
-        CU(cudaMemsetAsync(tb.llpart, 0, (size_t)Q * 8, ctx->stream));
+        CU(cudaMemsetAsync(tb.llpart, 0, (size_t)Q * 16, ctx->stream));
         CHECK(prof_begin(ctx));
         KL(launch_em_tc(ctx->stream, X, n, D, K, mu, ctx->w2(), ctx->c2(), tb, Q, ctx->tc_flush, &ctx->result()->status));
         CHECK(prof_end(ctx));
-        KL(launch_reduce_ll(ctx->stream, tb.llpart, Q, &ctx->result()->ll[slot], true));
+        KL(launch_reduce_ll(ctx->stream, tb.llpart, 2 * Q, &ctx->result()->ll[slot], true));
         KL(launch_reduce_tc(ctx->stream, D, K, Q, tb, Nk, S1, S2, true));
         return GMM_OK;
     }

@@ -65,6 +65,10 @@ int gmm_set_path(gmm_ctx* ctx, int path);
  * 22-bit split resolves, e.g. a component collapsed onto one point) have their competitive logits recomputed
  * exactly inside the kernel. */
 int gmm_tensor_path_supports(int D, int K);
+/* The path GMM_PATH_AUTO picks for shape (D, K): the tensor-core path when it is supported and the shape fills at
+ * least half of a 128-component MMA tile (K >= 64, D >= 8); otherwise the FP32 path, which is both faster and more
+ * accurate for small mixtures. */
+int gmm_auto_path(int D, int K);
 /* The path (GMM_PATH_FP32 or GMM_PATH_TENSOR) the most recent compute call actually ran. */
 int gmm_last_path(const gmm_ctx* ctx);
 

@@ -37,7 +37,7 @@ constexpr int NTHREADS = 416;          // 2 softmax warpgroups (even / odd tiles
 constexpr int MMA_WARP = 12;
 constexpr float RSCALE = TC_RSCALE;
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
-constexpr float ILL_ABS = 1000.f;
+constexpr float ILL_MARGIN = 40.f;     // log2 units: a logit more than this below the best one is negligible (2^-40)
 
 // shared memory map (offsets from a 1024-byte aligned base)
 constexpr int SM_PLO = 0;                       // 65536
@@ -49,14 +49,17 @@ constexpr int SM_GATHER = SM_MISC;              // 2 groups x 4 warps x 64 float
 constexpr int SM_WS = SM_GATHER + 2048;         // 2 groups x 4 warps x 64 float2    4096
 constexpr int SM_FAC = SM_WS + 4096;            // 2 groups x 4 warps x 64 floats    2048
 constexpr int SM_EXCH = SM_FAC + 2048;          // 2 bufs x 8 CTAs x 64 float2       8192
-constexpr int SM_SD = SM_EXCH + 8192;           // 128 floats                     512
+constexpr int SM_EXCH2 = SM_EXCH + 8192;        // 2 bufs x 8 CTAs x 64 floats       4096   (lower-bound exchange)
+constexpr int SM_LBW = SM_EXCH2 + 4096;         // 2 groups x 4 warps x 64 floats    2048
+constexpr int SM_LBG = SM_LBW + 2048;           // 2 groups x 64 floats               512
+constexpr int SM_SD = SM_LBG + 512;             // 128 floats                     512
 constexpr int SM_KAP = SM_SD + 512;             // 128 floats                     512
 constexpr int SM_LL = SM_KAP + 512;             // 2 x 64 doubles                1024
 constexpr int SM_BAR = SM_LL + 1024;             // barriers                       256
 constexpr int SM_END = SM_BAR + 256;
 constexpr int SMEM_BYTES = SM_END + 1024;       // + alignment slack
 
-enum { B_YFULL0 = 0, B_YFULL1, B_YEMPTY0, B_YEMPTY1, B_LFULL0, B_LFULL1, B_RREADY0, B_RREADY1, B_X0, B_X1, B_ACCFULL,
+enum { B_YFULL0 = 0, B_YFULL1, B_YEMPTY0, B_YEMPTY1, B_LFULL0, B_LFULL1, B_RREADY0, B_RREADY1, B_X0, B_X1, B_XL0, B_XL1, B_ACCFULL,
        B_ACCFREE, B_FINAL, B_COUNT };
 
 #ifdef FLASHGMM_DEBUG
@@ -138,6 +141,10 @@ __device__ __forceinline__ void st_remote_f2(uint32_t remote_addr, float a, floa
 __device__ __forceinline__ void st_async_f2(uint32_t remote_addr, float a, float b, uint32_t remote_bar) {
     asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.f32 [%0], {%1, %2}, [%3];"
                  ::"r"(remote_addr), "f"(a), "f"(b), "r"(remote_bar) : "memory");
+}
+__device__ __forceinline__ void st_async_f1(uint32_t remote_addr, float a, uint32_t remote_bar) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.f32 [%0], %1, [%2];"
+                 ::"r"(remote_addr), "f"(a), "r"(remote_bar) : "memory");
 }
 __device__ __forceinline__ void bar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
@@ -240,7 +247,8 @@ struct TcKernelParams {
     const float* ck;               // [CL*128]
     const float* sd;               // [128] per-dimension power-of-two data scale
     const float* kap;              // [128] per-dimension shift of the squares: Y = [s x | (s x)^2 + kap]
-    const float* illb;             // [CL*128] 0, or for an ill-conditioned component the log2 margin within which its logits are recomputed exactly
+    const float* illb;             // [CL*128] 0, or for an ill-conditioned component a bound E_k on the error of its approximate log2 z
+    const int* flags;              // [0] != 0 when some component is ill-conditioned (kernel-uniform protocol switch)
     const float* mu;               // [K][D] means (exact recomputation)
     const float* w2;               // [K][D] (log2 e / 2) / var
     const float* c2;               // [K] log2 e (log pi - 1/2 sum log(2 pi var))
@@ -281,6 +289,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
         bar_init(BAR(B_LFULL0), 1);    bar_init(BAR(B_LFULL1), 1);
         bar_init(BAR(B_RREADY0), 128); bar_init(BAR(B_RREADY1), 128);
         bar_init(BAR(B_X0), 1); bar_init(BAR(B_X1), 1);
+        bar_init(BAR(B_XL0), 1); bar_init(BAR(B_XL1), 1);
         bar_init(BAR(B_ACCFULL), 1);   bar_init(BAR(B_ACCFREE), 128);
         bar_init(BAR(B_FINAL), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -334,6 +343,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
         const float tk = p.tk[rank * 128 + kloc];
         const float ck = p.ck[rank * 128 + kloc];
         const float illb = p.illb[rank * 128 + kloc];
+        const bool any_ill = p.flags[0] != 0;
         float* gather = reinterpret_cast<float*>(smem + SM_GATHER) + warp * 64;
         float2* ws = reinterpret_cast<float2*>(smem + SM_WS) + grp * 256;      // [4][64] per group
         float* fac = reinterpret_cast<float*>(smem + SM_FAC) + grp * 256;      // [4][64] per group
@@ -373,64 +383,84 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                 for (int j = 0; j < 64; ++j) p.dbg[(size_t)(rank * 128 + kloc) * 64 + j] = l[j];
 #endif
             TOC(tk_, 16);
-            // warp-level max per point, all-gathered through shared memory
             float red[2];
-            warp_reduce_scatter<true>(l, red, lane);
-            reinterpret_cast<float2*>(gather)[lane] = make_float2(red[0], red[1]);
-            __syncwarp();
             // Ill-conditioned components (sum_d mu^2 / var too large for the 22-bit expanded form, e.g. a component
             // that collapsed onto a few points): wherever such a component is within reach of the warp's maximum for a
             // point, its logit is recomputed exactly with direct differences in fp32, the whole warp working on one
             // (component, point) pair at a time.  Rare by construction: a tight component is competitive for few points.
-            if (__any_sync(0xffffffffu, illb > 0.f)) {
-                uint32_t mlo = 0, mhi = 0;
+            // Ill-conditioned components (sum_d mu^2 / var too large for the 22-bit expanded form, e.g. a component
+            // collapsed onto a few points): their approximate logits carry an error of up to E_k.  A (component, point)
+            // pair can only matter if its upper bound l + E_k reaches the best LOWER bound max_k' (l - E_k') over ALL K
+            // components minus the 2^-40 margin, so the lower bounds are maximised over the cluster first (one extra
+            // exchange, only in launches that have such components).  Pairs that pass are recomputed exactly with
+            // direct differences in fp32, the whole warp working on one pair at a time; the rest are provably negligible.
+            if (any_ill) {
+                float* lbw = reinterpret_cast<float*>(smem + SM_LBW) + grp * 256;       // [4][64]
+                float* lbg = reinterpret_cast<float*>(smem + SM_LBG) + grp * 64;        // [64]
+                float* exch2 = reinterpret_cast<float*>(smem + SM_EXCH2);               // [2][8][64]
                 if (illb > 0.f) {
-                    // Two conditions: within `illb` of the warp's best logit for the point, and not absurdly far from the
-                    // component in absolute terms (log2 z - c_k = -log2e/2 * Mahalanobis^2 >= -ILL_ABS, about ten times the
-                    // expected D/2): the second one keeps ordinary points of other components, for which every
-                    // component of this warp is equally hopeless, out of the exact path.
-                    const float floor_abs = ck - ILL_ABS - illb;
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        if (l[j] >= floor_abs && j < nvalid && l[j] >= gather[j] - illb) mlo |= 1u << j;
-                        if (l[32 + j] >= floor_abs && 32 + j < nvalid && l[32 + j] >= gather[32 + j] - illb) mhi |= 1u << j;
-                    }
+                    for (int j = 0; j < 64; ++j) l[j] -= illb;
                 }
-                bool fixed_any = false;
-                const int kglob = (int)rank * 128 + kloc;
-                for (;;) {
-                    const uint32_t ballot = __ballot_sync(0xffffffffu, (mlo | mhi) != 0u);
-                    if (ballot == 0u) break;
-                    const int src = __ffs(ballot) - 1;
-                    int j = mlo ? (__ffs(mlo) - 1) : (32 + __ffs(mhi) - 1);
-                    j = __shfl_sync(0xffffffffu, j, src);
-                    const int kk = __shfl_sync(0xffffffffu, kglob, src);
-                    const float* xr = p.X + (row0 + j) * p.D;
-                    const float* mr = p.mu + (size_t)kk * p.D;
-                    const float* wr = p.w2 + (size_t)kk * p.D;
-                    float q = 0.f;
-                    for (int d = lane; d < p.D; d += 32) {
-                        const float diff = __ldg(xr + d) - __ldg(mr + d);
-                        q = fmaf(diff * diff, __ldg(wr + d), q);
-                    }
+                warp_reduce_scatter<true>(l, red, lane);
+                if (illb > 0.f) {
 #pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
-                    const float val = __ldg(p.c2 + kk) - q;
-                    if (lane == src) {
-#pragma unroll
-                        for (int jj = 0; jj < 64; ++jj)
-                            if (jj == j) l[jj] = val;
-                        if (j < 32) mlo &= ~(1u << j); else mhi &= ~(1u << (j - 32));
-                    }
-                    fixed_any = true;
+                    for (int j = 0; j < 64; ++j) l[j] += illb;      // (restores l up to ulp(E_k): irrelevant next to E_k)
                 }
-                if (fixed_any) {
-                    __syncwarp();
-                    warp_reduce_scatter<true>(l, red, lane);
-                    reinterpret_cast<float2*>(gather)[lane] = make_float2(red[0], red[1]);
-                    __syncwarp();
+                reinterpret_cast<float2*>(lbw + wq * 64)[lane] = make_float2(red[0], red[1]);
+                named_bar_sync(7 + 2 * grp, 128);
+                if (gtid < 64) {
+                    const float m4 = fmaxf(fmaxf(lbw[gtid], lbw[64 + gtid]), fmaxf(lbw[128 + gtid], lbw[192 + gtid]));
+                    const uint32_t slot2 = smem_u32(&exch2[(s * 8 + rank) * 64 + gtid]);
+                    if (gtid == 0) bar_arrive_expect_tx(BAR(B_XL0 + s), (uint32_t)p.CL * 64u * 4u);
+                    for (int c = 0; c < p.CL; ++c) st_async_f1(map_to_cta(slot2, c), m4, map_to_cta(BAR(B_XL0 + s), c));
+                    if (!bar_wait(BAR(B_XL0 + s), ph, abort_flag, p.status, false)) alive = false;
+                    float mg = -CUDART_INF_F;
+                    for (int c = 0; c < p.CL; ++c) mg = fmaxf(mg, exch2[(s * 8 + c) * 64 + gtid]);
+                    lbg[gtid] = mg;
+                }
+                named_bar_sync(8 + 2 * grp, 128);
+                if (__any_sync(0xffffffffu, illb > 0.f)) {
+                    const int kglob = (int)rank * 128 + kloc;
+                    uint32_t mlo = 0, mhi = 0;
+                    if (illb > 0.f) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            if (j < nvalid && l[j] + illb >= lbg[j] - ILL_MARGIN) mlo |= 1u << j;
+                            if (32 + j < nvalid && l[32 + j] + illb >= lbg[32 + j] - ILL_MARGIN) mhi |= 1u << j;
+                        }
+                    }
+                    for (;;) {
+                        const uint32_t ballot = __ballot_sync(0xffffffffu, (mlo | mhi) != 0u);
+                        if (ballot == 0u) break;
+                        const int src = __ffs(ballot) - 1;
+                        int j = mlo ? (__ffs(mlo) - 1) : (32 + __ffs(mhi) - 1);
+                        j = __shfl_sync(0xffffffffu, j, src);
+                        const int kk = __shfl_sync(0xffffffffu, kglob, src);
+                        const float* xr = p.X + (row0 + j) * p.D;
+                        const float* mr = p.mu + (size_t)kk * p.D;
+                        const float* wr = p.w2 + (size_t)kk * p.D;
+                        float q = 0.f;
+                        for (int d = lane; d < p.D; d += 32) {
+                            const float diff = __ldg(xr + d) - __ldg(mr + d);
+                            q = fmaf(diff * diff, __ldg(wr + d), q);
+                        }
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
+                        const float val = __ldg(p.c2 + kk) - q;
+                        if (lane == src) {
+#pragma unroll
+                            for (int jj = 0; jj < 64; ++jj)
+                                if (jj == j) l[jj] = val;
+                            if (j < 32) mlo &= ~(1u << j); else mhi &= ~(1u << (j - 32));
+                        }
+                    }
                 }
             }
+            // warp-level max per point, all-gathered through shared memory
+            warp_reduce_scatter<true>(l, red, lane);
+            reinterpret_cast<float2*>(gather)[lane] = make_float2(red[0], red[1]);
+            __syncwarp();
             TOC(tk_, 17);
             const float mw_mine0 = red[0], mw_mine1 = red[1];
 #pragma unroll
@@ -754,7 +784,7 @@ __global__ void __launch_bounds__(128) tc_prepare_kernel(int D, int K, const flo
                                                          uint32_t* __restrict__ phi_img,
                                                          unsigned char* __restrict__ plo_img, float* __restrict__ tk,
                                                          float* __restrict__ ck, float* __restrict__ illb, float cond_limit,
-                                                         int* __restrict__ status) {
+                                                         int* __restrict__ flags) {
     const int k = blockIdx.x, d = threadIdx.x;
     const int slice = k >> 7, row = k & 127;
     __shared__ double red_max[128], red_c[128], red_cond[128], red_k[128];
@@ -818,8 +848,8 @@ __global__ void __launch_bounds__(128) tc_prepare_kernel(int D, int K, const flo
         const double cond = red_cond[0] * 2.384185791015625e-07;
         float margin = 0.f;
         if (k < K && cond > (double)cond_limit) {
-            margin = (float)fmin(40.0 + 8.0 * cond, 1e30);
-            atomicOr(status, ST_ILLCOND);
+            margin = (float)fmin(8.0 * cond, 1e30);       // E_k: error bound of the approximate log2 z (8 x the estimate)
+            atomicOr(flags, 1);
         }
         illb[k] = margin;
     }
@@ -895,10 +925,13 @@ size_t tc_scratch_bytes(int D, int K) {
 cudaError_t launch_prepare_tc(cudaStream_t s, int D, int K, const float* pi, const float* mu, const float* var,
                               const TcBuffers& tb, float cond_limit, int* status) {
     const TcPlan pl = tc_plan(D, K, 148);
+    (void)status;
+    cudaError_t e0 = cudaMemsetAsync(tb.flags, 0, sizeof(int), s);
+    if (e0 != cudaSuccess) return e0;
     tc_scale_kernel<<<1, 128, 0, s>>>(D, K, pi, mu, var, tb.sd, tb.kap);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    tc_prepare_kernel<<<pl.Kpad, 128, 0, s>>>(D, K, pi, mu, var, tb.sd, tb.kap, tb.phi_img, tb.plo_img, tb.tk, tb.ck, tb.illb, cond_limit, status);
+    tc_prepare_kernel<<<pl.Kpad, 128, 0, s>>>(D, K, pi, mu, var, tb.sd, tb.kap, tb.phi_img, tb.plo_img, tb.tk, tb.ck, tb.illb, cond_limit, tb.flags);
     return cudaGetLastError();
 }
 
@@ -909,7 +942,7 @@ cudaError_t launch_em_tc(cudaStream_t s, const float* X, int64_t n, int D, int K
     p.X = X; p.n = n; p.D = D; p.K = K; p.CL = pl.CL; p.Q = Q; p.n_ks = pl.n_ks;
     p.flush = (flush_tiles < 2) ? 2 : (flush_tiles & ~1);
     p.phi_img = tb.phi_img; p.plo_img = tb.plo_img; p.tk = tb.tk; p.ck = tb.ck; p.sd = tb.sd; p.kap = tb.kap;
-    p.illb = tb.illb; p.mu = mu; p.w2 = w2; p.c2 = c2;
+    p.illb = tb.illb; p.flags = tb.flags; p.mu = mu; p.w2 = w2; p.c2 = c2;
     p.partial = tb.partial; p.llpart = tb.llpart; p.status = status;
 #ifdef FLASHGMM_DEBUG
     p.dbg = g_tc_debug;

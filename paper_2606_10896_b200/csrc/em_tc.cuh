@@ -26,6 +26,7 @@ struct TcBuffers {
     float* sd;
     float* kap;
     float* illb;
+    int* flags;
     double* partial;
     double* llpart;
 };

@@ -28,7 +28,7 @@ inline size_t align256(size_t b) { return (b + 255) & ~(size_t)255; }
 
 struct ScratchLayout {
     size_t w2, c2, partials, logZ2, llpart, result, stats, total;
-    size_t tc_phi, tc_plo, tc_tk, tc_ck, tc_sd, tc_kap, tc_illb, tc_partial, tc_llpart, tc_partial_bytes;
+    size_t tc_phi, tc_plo, tc_tk, tc_ck, tc_sd, tc_kap, tc_illb, tc_flags, tc_partial, tc_llpart, tc_partial_bytes;
     bool tc;
 };
 
@@ -45,7 +45,7 @@ ScratchLayout scratch_layout(int D, int K) {
     L.result = take(sizeof(DevResult));
     L.stats = take(((size_t)K + 2 * KD) * 8);
     L.tc = tc_supports(D, K);
-    L.tc_phi = L.tc_plo = L.tc_tk = L.tc_ck = L.tc_sd = L.tc_kap = L.tc_illb = L.tc_partial = L.tc_llpart = 0;
+    L.tc_phi = L.tc_plo = L.tc_tk = L.tc_ck = L.tc_sd = L.tc_kap = L.tc_illb = L.tc_flags = L.tc_partial = L.tc_llpart = 0;
     L.tc_partial_bytes = 0;
     if (L.tc) {
         const TcPlan pl = tc_plan(D, K, 160);       // an upper bound on the number of clusters
@@ -56,6 +56,7 @@ ScratchLayout scratch_layout(int D, int K) {
         L.tc_sd = take(128 * 4);
         L.tc_kap = take(128 * 4);
         L.tc_illb = take((size_t)pl.Kpad * 4);
+        L.tc_flags = take(16);
         L.tc_partial_bytes = (size_t)pl.Q * pl.Kpad * TC_PCOLS * 8;
         L.tc_partial = take(L.tc_partial_bytes);
         L.tc_llpart = take((size_t)pl.Q * 16);
@@ -77,7 +78,8 @@ struct gmm_ctx {
     int capD = 0, capK = 0;
     ScratchLayout lay{};
     int tc_Q = 0;              // resident clusters of the tensor-path kernel for (capD, capK)
-    float tc_cond_limit = 3e-3f;
+    float tc_cond_limit = -1.f;      // < 0: automatic, tc_cond_scale * sqrt(N / K)
+    float tc_cond_scale = 1.5e-4f;
     int tc_flush = TC_FLUSH;
     // host-streaming path
     cudaStream_t copy_stream = nullptr;
@@ -111,6 +113,7 @@ struct gmm_ctx {
         b.sd = reinterpret_cast<float*>(scratch + lay.tc_sd);
         b.kap = reinterpret_cast<float*>(scratch + lay.tc_kap);
         b.illb = reinterpret_cast<float*>(scratch + lay.tc_illb);
+        b.flags = reinterpret_cast<int*>(scratch + lay.tc_flags);
         b.partial = reinterpret_cast<double*>(scratch + lay.tc_partial);
         b.llpart = reinterpret_cast<double*>(scratch + lay.tc_llpart);
         return b;
@@ -228,17 +231,24 @@ int prof_end(gmm_ctx* ctx) {
 
 // Derived per-component constants for both paths; validates the parameters into the status word.  Then picks the
 // path: the tensor-core path whenever the shape allows it (ill-conditioned components are handled inside its kernel).
-int prepare_and_choose(gmm_ctx* ctx, int D, int K, const float* pi, const float* mu, const float* var, int* path) {
+int prepare_and_choose(gmm_ctx* ctx, int64_t N, int D, int K, const float* pi, const float* mu, const float* var,
+                       int* path) {
     CU(cudaMemsetAsync(&ctx->result()->status, 0, sizeof(int), ctx->stream));
     KL(launch_prepare_fp32(ctx->stream, D, K, pi, mu, var, ctx->w2(), ctx->c2(), &ctx->result()->status));
     const bool tc_ok = ctx->lay.tc && ctx->tc_Q >= 1;
+    const bool tc_auto = tc_ok && gmm_auto_path(D, K) == GMM_PATH_TENSOR;
     if (ctx->path == GMM_PATH_TENSOR && !tc_ok)
         return fail(ctx, GMM_EUNSUPPORTED, "the tensor-core path needs D <= 128 and K <= 1024 (got D=%d K=%d)", D, K);
-    if (ctx->path == GMM_PATH_FP32 || !tc_ok) {
+    if (ctx->path == GMM_PATH_FP32 || !tc_ok || (ctx->path == GMM_PATH_AUTO && !tc_auto)) {
         *path = GMM_PATH_FP32;
         return GMM_OK;
     }
-    KL(launch_prepare_tc(ctx->stream, D, K, pi, mu, var, ctx->tc(), ctx->tc_cond_limit, &ctx->result()->status));
+    // Components whose estimated logit error exceeds the limit get their competitive logits recomputed exactly.  The
+    // error a responsibility may carry shrinks with the number of points that average it out, so the limit follows
+    // sqrt(points per component): parameter errors stay below 1e-4 of the data scale at any N / K.
+    float limit = ctx->tc_cond_limit;
+    if (limit < 0.f) limit = ctx->tc_cond_scale * std::sqrt((float)((double)N / (double)K));
+    KL(launch_prepare_tc(ctx->stream, D, K, pi, mu, var, ctx->tc(), limit, &ctx->result()->status));
     ctx->launches++;   // launch_prepare_tc enqueues two kernels
     *path = GMM_PATH_TENSOR;
     return GMM_OK;
@@ -377,7 +387,7 @@ int gmm_em_step(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const flo
     DeviceGuard g(ctx->device);
     int path;
     CHECK(ensure_scratch(ctx, D, K));
-    CHECK(prepare_and_choose(ctx, D, K, pi, mu, var, &path));
+    CHECK(prepare_and_choose(ctx, N, D, K, pi, mu, var, &path));
     CHECK(zero_stats(ctx, D, K, Nk, S1, S2, 0));
     CHECK(accumulate_points(ctx, path, X, N, D, K, mu, Nk, S1, S2, 0));
     ctx->last_path = path;
@@ -420,7 +430,7 @@ int gmm_fit(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, float* pi, fl
     int t = 0;
     for (; t < iters; ++t) {
         const int slot = t % LL_SLOTS;
-        CHECK(prepare_and_choose(ctx, D, K, pi, mu, var, &path));
+        CHECK(prepare_and_choose(ctx, N, D, K, pi, mu, var, &path));
         CHECK(zero_stats(ctx, D, K, Nk, S1, S2, slot));
         CHECK(accumulate_points(ctx, path, X, N, D, K, mu, Nk, S1, S2, slot));
         KL(launch_finalize(ctx->stream, N, D, K, Nk, S1, S2, var_floor, pi, mu, var));
@@ -494,7 +504,7 @@ int gmm_em_step_host(gmm_ctx* ctx, const float* X_host, int64_t N, int D, int K,
     double* Nk = ctx->stats();
     double* S1 = Nk + K;
     double* S2 = S1 + KD;
-    CHECK(prepare_and_choose(ctx, D, K, pi, mu, var, &path));
+    CHECK(prepare_and_choose(ctx, N, D, K, pi, mu, var, &path));
     CHECK(zero_stats(ctx, D, K, Nk, S1, S2, 0));
     const int64_t rows_per_chunk = (int64_t)(STAGE_BYTES / ((size_t)D * 4));
     if (rows_per_chunk < 1) return fail(ctx, GMM_EINVAL, "D too large for the staging buffer");
@@ -539,6 +549,8 @@ int gmm_assign_topm(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const
 }
 
 int gmm_tensor_path_supports(int D, int K) { return tc_supports(D, K) ? 1 : 0; }
+
+int gmm_auto_path(int D, int K) { return (tc_supports(D, K) && K >= 64 && D >= 8) ? GMM_PATH_TENSOR : GMM_PATH_FP32; }
 
 size_t gmm_scratch_bytes(int D, int K) {
     if (D < 1 || K < 1) return 0;

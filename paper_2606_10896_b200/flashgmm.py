@@ -27,6 +27,7 @@ EXPORTS = {
     "gmm_set_path": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int]),
     "gmm_last_path": (ctypes.c_int, [ctypes.c_void_p]),
     "gmm_tensor_path_supports": (ctypes.c_int, [ctypes.c_int, ctypes.c_int]),
+    "gmm_auto_path": (ctypes.c_int, [ctypes.c_int, ctypes.c_int]),
     "gmm_em_step": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_int,
                                    ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                    ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
@@ -85,6 +86,10 @@ class GmmError(RuntimeError):
 
 def tensor_path_supports(D: int, K: int) -> bool:
     return bool(lib.gmm_tensor_path_supports(int(D), int(K)))
+
+
+def gmm_auto_path(D: int, K: int) -> int:
+    return int(lib.gmm_auto_path(int(D), int(K)))
 
 
 def gmm_scratch_bytes(D: int, K: int) -> int:

@@ -252,7 +252,7 @@ struct TcKernelParams {
     const float* mu;               // [K][D] means (exact recomputation)
     const float* w2;               // [K][D] (log2 e / 2) / var
     const float* c2;               // [K] log2 e (log pi - 1/2 sum log(2 pi var))
-    double* partial;               // [Q][CL*128][TC_PCOLS]  (+=)
+    double* partial;               // [Q][TC_PCOLS][CL*128]  (+=)
     double* llpart;                // [Q]
     int* status;
 #ifdef FLASHGMM_DEBUG
@@ -350,7 +350,10 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
         float2* exch = reinterpret_cast<float2*>(smem + SM_EXCH);      // [2][8][64]
         float nk_acc = 0.f;
         double ll_acc = 0.0;
-        double* prow = p.partial + ((size_t)cluster_id * (p.CL * 128) + rank * 128 + kloc) * TC_PCOLS;
+        // partial layout [cluster][column][component]: the 32 lanes of a warp touch 32 consecutive doubles; every address
+        // belongs to exactly one thread of the grid, so the reductions below are deterministic
+        const size_t pstride = (size_t)p.CL * 128;
+        double* prow = p.partial + (size_t)cluster_id * TC_PCOLS * pstride + rank * 128 + kloc;
         bool alive = true;
 
         // Softmax threads leave the loop only at the uniform decision point after named barrier 2: a thread that
@@ -567,7 +570,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                     tmem_ld32(T_ACC + lane_addr + c0, v);
                     tmem_wait_ld();
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) prow[c0 + j] += (double)__uint_as_float(v[j]);
+                    for (int j = 0; j < 32; ++j) atomicAdd(prow + (size_t)(c0 + j) * pstride, (double)__uint_as_float(v[j]));
                 }
                 fence_before();
                 bar_arrive(BAR(B_ACCFREE));
@@ -575,7 +578,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
             }
             // N_k of this group's tiles has its own column, flushed on the group's own cadence
             if ((((i >> 1) + 1) % 32) == 0 || i + 2 >= ntl) {
-                prow[256 + grp] += (double)nk_acc;
+                atomicAdd(prow + (size_t)(256 + grp) * pstride, (double)nk_acc);
                 nk_acc = 0.f;
             }
         }
@@ -876,13 +879,13 @@ __global__ void tc_reduce_kernel(int D, int K, int Kpad, int Q, const double* __
         col = 16 * (d >> 3) + (d & 7) + 8; unscale /= (double)sd[d] * (double)sd[d]; dst = S2 + j;
     }
     double s = 0.0;
-    for (int q = 0; q < Q; ++q) s += partial[((size_t)q * Kpad + k) * TC_PCOLS + col];
+    for (int q = 0; q < Q; ++q) s += partial[((size_t)q * TC_PCOLS + col) * Kpad + k];
     if (e < (size_t)K)
-        for (int q = 0; q < Q; ++q) s += partial[((size_t)q * Kpad + k) * TC_PCOLS + 257];
+        for (int q = 0; q < Q; ++q) s += partial[((size_t)q * TC_PCOLS + 257) * Kpad + k];
     if (e >= K + KD) {          // squares were accumulated as (s x)^2 + kap: take kap * N_k out again
         const int d = (int)((e - K - KD) % D);
         double nk = 0.0;
-        for (int q = 0; q < Q; ++q) nk += partial[((size_t)q * Kpad + k) * TC_PCOLS + 256] + partial[((size_t)q * Kpad + k) * TC_PCOLS + 257];
+        for (int q = 0; q < Q; ++q) nk += partial[((size_t)q * TC_PCOLS + 256) * Kpad + k] + partial[((size_t)q * TC_PCOLS + 257) * Kpad + k];
         s -= (double)kap[d] * nk;
     }
     s *= unscale;

@@ -4,8 +4,8 @@
 //   E-step   L[k, i] = sum_c P[k, c] * Y[i, c]         P = per-component coefficients (a = log2e mu/var, b = -log2e/(2 var)),
 //                                                      Y = [x | x^2], contraction length 2 * 128 padded dimensions
 //   log2 z_ik = t_k * L[k, i] + c_k                     (row scale t_k, constant c_k = log2e (log pi_k - 1/2 sum_d (mu^2/var + log 2 pi var)))
-//   log-sum-exp over ALL K components of a point        (warp butterflies, then one (max, sum) exchange per tile between the CTAs of a cluster
-//                                                        through distributed shared memory: each CTA owns 128 components)
+//   log-sum-exp over ALL K components of a point        (warp butterflies, then one (max, sum) exchange per tile between the ceil(K/128) CTAs of a
+//                                                        group through tagged slots in global memory (L2): each CTA owns 128 components)
 //   r_ik = 2^(log2 z_ik - log2 Z_i)                     on chip only: written back into TMEM as the A operand of the M-step
 //   M-step   S[k, c] += sum_i r_ik * Y[i, c]            accumulators stationary in TMEM for the CTA's whole life
 // Precision: every operand is split into two fp16 values (hi + lo, 22 bits).  E-step = P_hi Y_hi + P_hi Y_lo + P_lo Y_hi,
@@ -48,9 +48,7 @@ constexpr int SM_MISC = SM_Y + 2 * SM_YSTAGE;   // 196608
 constexpr int SM_GATHER = SM_MISC;              // 2 groups x 4 warps x 64 floats    2048
 constexpr int SM_WS = SM_GATHER + 2048;         // 2 groups x 4 warps x 64 float2    4096
 constexpr int SM_FAC = SM_WS + 4096;            // 2 groups x 4 warps x 64 floats    2048
-constexpr int SM_EXCH = SM_FAC + 2048;          // 2 bufs x 8 CTAs x 64 float2       8192
-constexpr int SM_EXCH2 = SM_EXCH + 8192;        // 2 bufs x 8 CTAs x 64 floats       4096   (lower-bound exchange)
-constexpr int SM_LBW = SM_EXCH2 + 4096;         // 2 groups x 4 warps x 64 floats    2048
+constexpr int SM_LBW = SM_FAC + 2048;           // 2 groups x 4 warps x 64 floats    2048
 constexpr int SM_LBG = SM_LBW + 2048;           // 2 groups x 64 floats               512
 constexpr int SM_SD = SM_LBG + 512;             // 128 floats                     512
 constexpr int SM_KAP = SM_SD + 512;             // 128 floats                     512
@@ -59,7 +57,7 @@ constexpr int SM_BAR = SM_LL + 1024;             // barriers                    
 constexpr int SM_END = SM_BAR + 256;
 constexpr int SMEM_BYTES = SM_END + 1024;       // + alignment slack
 
-enum { B_YFULL0 = 0, B_YFULL1, B_YEMPTY0, B_YEMPTY1, B_LFULL0, B_LFULL1, B_RREADY0, B_RREADY1, B_X0, B_X1, B_XL0, B_XL1, B_ACCFULL,
+enum { B_YFULL0 = 0, B_YFULL1, B_YEMPTY0, B_YEMPTY1, B_LFULL0, B_LFULL1, B_RREADY0, B_RREADY1, B_ACCFULL,
        B_ACCFREE, B_FINAL, B_COUNT };
 
 #ifdef FLASHGMM_DEBUG
@@ -126,38 +124,19 @@ __device__ __forceinline__ void bar_init(uint32_t bar, uint32_t count) {
 __device__ __forceinline__ void bar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void bar_arrive_remote(uint32_t remote_bar) {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote_bar) : "memory");
+// ---- exchange between the CTAs of a group through global memory (L2).  A slot is two 64-bit words {value, tag}: each
+//      word is written and read as one unit, so a reader that sees the expected tag in both words has both values.
+//      Slots form a ring of 4 per (group, source CTA): a CTA writes tile i+4 only after it has finished tile i+2, which
+//      needed every peer's tile-(i+2) slot, which that peer wrote after it had read all slots of tile i.
+struct __align__(16) XSlot { float a; uint32_t ta; float b; uint32_t tb; };
+__device__ __forceinline__ void xslot_write(XSlot* q, float a, float b, uint32_t tag) {
+    asm volatile("st.relaxed.gpu.global.v4.b32 [%0], {%1, %2, %3, %4};"
+                 ::"l"(q), "r"(__float_as_uint(a)), "r"(tag), "r"(__float_as_uint(b)), "r"(tag) : "memory");
 }
-__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t cta_rank) {
-    uint32_t r;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(cta_rank));
-    return r;
+__device__ __forceinline__ void xslot_load(const XSlot* q, uint32_t (&v)[4]) {
+    asm volatile("ld.relaxed.gpu.global.v4.b32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]) : "l"(q) : "memory");
 }
-__device__ __forceinline__ void st_remote_f2(uint32_t remote_addr, float a, float b) {
-    asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(remote_addr), "f"(a), "f"(b) : "memory");
-}
-// Remote 8-byte store that signals the destination CTA's mbarrier with its byte count (no release round trip).
-__device__ __forceinline__ void st_async_f2(uint32_t remote_addr, float a, float b, uint32_t remote_bar) {
-    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.f32 [%0], {%1, %2}, [%3];"
-                 ::"r"(remote_addr), "f"(a), "f"(b), "r"(remote_bar) : "memory");
-}
-__device__ __forceinline__ void st_async_f1(uint32_t remote_addr, float a, uint32_t remote_bar) {
-    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.f32 [%0], %1, [%2];"
-                 ::"r"(remote_addr), "f"(a), "r"(remote_bar) : "memory");
-}
-__device__ __forceinline__ void bar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ uint32_t cluster_rank() {
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-__device__ __forceinline__ void cluster_sync_all() {
-    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-
 // Bounded wait on an mbarrier phase.  Returns false on abort/timeout (and raises the abort flag).
 __device__ __forceinline__ bool bar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, bool cluster_scope) {
     unsigned long long t0 = 0;
@@ -170,6 +149,26 @@ __device__ __forceinline__ bool bar_wait(uint32_t bar, uint32_t parity, volatile
             asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
                          : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
         if (ok) return true;
+        if (*abort_flag) return false;
+        if ((it & 63) == 63) {
+            const unsigned long long now = gtime();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > WAIT_LIMIT_NS) {
+                *abort_flag = 1;
+                atomicOr(status, ST_TIMEOUT);
+                return false;
+            }
+        }
+    }
+}
+
+// Bounded poll of an exchange slot until both tags match.
+__device__ __forceinline__ bool xslot_wait(const XSlot* q, uint32_t tag, float& a, float& b, volatile int* abort_flag, int* status) {
+    unsigned long long t0 = 0;
+    for (int it = 0;; ++it) {
+        uint32_t v[4];
+        xslot_load(q, v);
+        if (v[1] == tag && v[3] == tag) { a = __uint_as_float(v[0]); b = __uint_as_float(v[2]); return true; }
         if (*abort_flag) return false;
         if ((it & 63) == 63) {
             const unsigned long long now = gtime();
@@ -253,7 +252,9 @@ struct TcKernelParams {
     const float* w2;               // [K][D] (log2 e / 2) / var
     const float* c2;               // [K] log2 e (log pi - 1/2 sum log(2 pi var))
     double* partial;               // [Q][TC_PCOLS][CL*128]  (+=)
-    double* llpart;                // [Q]
+    double* llpart;                // [2 Q]
+    XSlot* xg;                     // [Q][4][CL][64] exchange slots (zeroed before every launch)
+    XSlot* xl;                     // [Q][4][CL][64] lower-bound exchange slots
     int* status;
 #ifdef FLASHGMM_DEBUG
     float* dbg;      // [Kpad][64] log2 z of the first tile
@@ -270,8 +271,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
     volatile int* abort_flag = &abort_s;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const uint32_t rank = (p.CL > 1) ? cluster_rank() : 0;
-    const int cluster_id = blockIdx.x / p.CL;
+    const uint32_t rank = blockIdx.x % p.CL;          // slice of 128 components within the group
+    const int cluster_id = blockIdx.x / p.CL;          // group index: a group of CL CTAs covers all K components of its tiles
     const int64_t ntiles = (p.n + BN - 1) / BN;
     const int64_t ntl = (cluster_id < ntiles) ? (ntiles - cluster_id + p.Q - 1) / p.Q : 0;   // tiles of this cluster
 
@@ -288,8 +289,6 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
         bar_init(BAR(B_YEMPTY0), 1);   bar_init(BAR(B_YEMPTY1), 1);
         bar_init(BAR(B_LFULL0), 1);    bar_init(BAR(B_LFULL1), 1);
         bar_init(BAR(B_RREADY0), 128); bar_init(BAR(B_RREADY1), 128);
-        bar_init(BAR(B_X0), 1); bar_init(BAR(B_X1), 1);
-        bar_init(BAR(B_XL0), 1); bar_init(BAR(B_XL1), 1);
         bar_init(BAR(B_ACCFULL), 1);   bar_init(BAR(B_ACCFREE), 128);
         bar_init(BAR(B_FINAL), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -331,7 +330,6 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
     fence_before();
     __syncthreads();
     fence_after();
-    if (p.CL > 1) cluster_sync_all();      // peers' barriers are initialised before anyone sends to them
 
     if (warp < 8) {
         // =========================== softmax warps ===========================
@@ -347,7 +345,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
         float* gather = reinterpret_cast<float*>(smem + SM_GATHER) + warp * 64;
         float2* ws = reinterpret_cast<float2*>(smem + SM_WS) + grp * 256;      // [4][64] per group
         float* fac = reinterpret_cast<float*>(smem + SM_FAC) + grp * 256;      // [4][64] per group
-        float2* exch = reinterpret_cast<float2*>(smem + SM_EXCH);      // [2][8][64]
+        XSlot* xg = p.xg + (size_t)cluster_id * 4 * p.CL * 64;             // [4][CL][64] ring of exchange slots
+        XSlot* xl = p.xl + (size_t)cluster_id * 4 * p.CL * 64;             // same, for the lower-bound exchange
         float nk_acc = 0.f;
         double ll_acc = 0.0;
         // partial layout [cluster][column][component]: the 32 lanes of a warp touch 32 consecutive doubles; every address
@@ -400,7 +399,6 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
             if (any_ill) {
                 float* lbw = reinterpret_cast<float*>(smem + SM_LBW) + grp * 256;       // [4][64]
                 float* lbg = reinterpret_cast<float*>(smem + SM_LBG) + grp * 64;        // [64]
-                float* exch2 = reinterpret_cast<float*>(smem + SM_EXCH2);               // [2][8][64]
                 if (illb > 0.f) {
 #pragma unroll
                     for (int j = 0; j < 64; ++j) l[j] -= illb;
@@ -414,12 +412,15 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                 named_bar_sync(7 + 2 * grp, 128);
                 if (gtid < 64) {
                     const float m4 = fmaxf(fmaxf(lbw[gtid], lbw[64 + gtid]), fmaxf(lbw[128 + gtid], lbw[192 + gtid]));
-                    const uint32_t slot2 = smem_u32(&exch2[(s * 8 + rank) * 64 + gtid]);
-                    if (gtid == 0) bar_arrive_expect_tx(BAR(B_XL0 + s), (uint32_t)p.CL * 64u * 4u);
-                    for (int c = 0; c < p.CL; ++c) st_async_f1(map_to_cta(slot2, c), m4, map_to_cta(BAR(B_XL0 + s), c));
-                    if (!bar_wait(BAR(B_XL0 + s), ph, abort_flag, p.status, false)) alive = false;
+                    const uint32_t tag = (uint32_t)(i + 1);
+                    XSlot* ring = xl + (size_t)(i & 3) * p.CL * 64;
+                    xslot_write(ring + rank * 64 + gtid, m4, 0.f, tag);
                     float mg = -CUDART_INF_F;
-                    for (int c = 0; c < p.CL; ++c) mg = fmaxf(mg, exch2[(s * 8 + c) * 64 + gtid]);
+                    for (int c = 0; c < p.CL; ++c) {
+                        float a = -CUDART_INF_F, b = 0.f;
+                        if (!xslot_wait(ring + c * 64 + gtid, tag, a, b, abort_flag, p.status)) alive = false;
+                        mg = fmaxf(mg, a);
+                    }
                     lbg[gtid] = mg;
                 }
                 named_bar_sync(8 + 2 * grp, 128);
@@ -497,20 +498,22 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
 #pragma unroll
                 for (int w = 0; w < 4; ++w)       // a warp whose lanes are all padded / zero-weight has m_w = -inf: skip it
                     sc += (w4[w].x == -CUDART_INF_F) ? 0.f : w4[w].y * fast_ex2(w4[w].x - mc_safe);
-                // send (m, s) of this CTA's 128 components to every CTA of the cluster (including this one)
-                const uint32_t slot = smem_u32(&exch[(s * 8 + rank) * 64 + pt]);
-                if (pt == 0) bar_arrive_expect_tx(BAR(B_X0 + s), (uint32_t)p.CL * 64u * 8u);   // this tile's incoming bytes
-                for (int c = 0; c < p.CL; ++c) st_async_f2(map_to_cta(slot, c), mc, sc, map_to_cta(BAR(B_X0 + s), c));
+                // publish (m, s) of this CTA's 128 components, then collect the group's
+                const uint32_t tag = (uint32_t)(i + 1);
+                XSlot* ring = xg + (size_t)(i & 3) * p.CL * 64;
+                xslot_write(ring + rank * 64 + pt, mc, sc, tag);
                 TOC(tk_, 3);
-                if (!bar_wait(BAR(B_X0 + s), ph, abort_flag, p.status, false)) alive = false;
-                TOC(tk_, 4);
                 float mi = -CUDART_INF_F;
                 float2 e[8];
 #pragma unroll
                 for (int c = 0; c < 8; ++c) {
-                    e[c] = (c < p.CL) ? exch[(s * 8 + c) * 64 + pt] : make_float2(-CUDART_INF_F, 0.f);
+                    e[c] = make_float2(-CUDART_INF_F, 0.f);
+                    if (c < p.CL) {
+                        if (!xslot_wait(ring + c * 64 + pt, tag, e[c].x, e[c].y, abort_flag, p.status)) alive = false;
+                    }
                     mi = fmaxf(mi, e[c].x);
                 }
+                TOC(tk_, 4);
                 const float mi_safe = (mi == -CUDART_INF_F) ? 0.f : mi;
                 float Z = 0.f;
 #pragma unroll
@@ -716,6 +719,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
             TOC(tm_, 15);
             return true;
         };
+        // Issue order per pair of tiles: E(a) E(b) M(a) M(b).  (The interleaved order M(i) E(i+2) M(i+1) ... was measured
+        // slower: it puts the Y-stage refill between every M and the following E on the tensor pipe's critical path.)
         for (int64_t i = 0; i < ntl && alive; i += 2) {
             const bool has2 = i + 1 < ntl;
             alive = issue_E(i);
@@ -740,7 +745,6 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
     // teardown: everybody meets, peers are done with this CTA's shared memory, TMEM is released
     fence_before();
     __syncthreads();
-    if (p.CL > 1) cluster_sync_all();
     if (warp == MMA_WARP) {
         fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512) : "memory");
@@ -755,28 +759,40 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
 // contraction as (s x)^2 + kap_d, which turns the monotonically growing partial sums sum_d w (mu x - x^2 / 2) ~ sum_d w mu^2 / 2
 // into a zero-mean walk sum_d w (mu^2 - kap) / 2 (several times smaller), and with it the error of the fp32 accumulation
 // in the tensor core.  The constant is given back exactly through c_k (E-step) and kap_d N_k (M-step).
-__global__ void tc_scale_kernel(int D, int K, const float* __restrict__ pi, const float* __restrict__ mu,
-                                const float* __restrict__ var, float* __restrict__ sd, float* __restrict__ kap) {
-    const int d = threadIdx.x;
-    float s = 1.f, kp = 0.f;
+__global__ void __launch_bounds__(128) tc_scale_kernel(int D, int K, const float* __restrict__ pi, const float* __restrict__ mu,
+                                                       const float* __restrict__ var, float* __restrict__ sd,
+                                                       float* __restrict__ kap) {
+    // one block per dimension (padded to 128); threads stride over the components, fixed-shape tree reduction
+    const int d = blockIdx.x, t = threadIdx.x;
+    __shared__ double r_acc[128], r_m[128], r_w[128];
+    double acc = 0.0, accm = 0.0, wsum = 0.0;
     if (d < D) {
-        double acc = 0.0, accm = 0.0, wsum = 0.0;
-        for (int k = 0; k < K; ++k) {
+        for (int k = t; k < K; k += 128) {
             const double w = (double)pi[k];
             const double m = (double)mu[(size_t)k * D + d];
             acc += w * (m * m + (double)var[(size_t)k * D + d]);
             accm += w * m * m;
             wsum += w;
         }
+    }
+    r_acc[t] = acc; r_m[t] = accm; r_w[t] = wsum;
+    __syncthreads();
+    for (int o = 64; o > 0; o >>= 1) {
+        if (t < o) { r_acc[t] += r_acc[t + o]; r_m[t] += r_m[t + o]; r_w[t] += r_w[t + o]; }
+        __syncthreads();
+    }
+    if (t == 0) {
+        float s = 1.f, kp = 0.f;
+        acc = r_acc[0]; accm = r_m[0]; wsum = r_w[0];
         if (wsum > 0.0) { acc /= wsum; accm /= wsum; }
-        if (acc > 0.0 && isfinite(acc)) {
+        if (d < D && acc > 0.0 && isfinite(acc)) {
             const double e = rint(0.5 * log2(acc));
             s = (float)exp2(-fmin(fmax(e, -60.0), 60.0));
             kp = (float)(accm * (double)s * (double)s);      // mean of mu^2 in scaled units
         }
+        sd[d] = s;
+        kap[d] = kp;
     }
-    sd[d] = s;
-    kap[d] = kp;
 }
 
 // One block (128 threads) per padded component: builds the P_hi TMEM image, the P_lo shared-memory image, t_k, c_k,
@@ -922,6 +938,7 @@ size_t tc_scratch_bytes(int D, int K) {
     b += (size_t)pl.Kpad * 4 * 2 + 512;                    // t_k, c_k, s_d
     b += (size_t)pl.Q * pl.Kpad * TC_PCOLS * 8;            // float64 partials
     b += (size_t)pl.Q * 16;
+    b += 2 * (size_t)pl.Q * 4 * pl.CL * 64 * 16;           // exchange slots
     return b + 8 * 256;
 }
 
@@ -931,7 +948,7 @@ cudaError_t launch_prepare_tc(cudaStream_t s, int D, int K, const float* pi, con
     (void)status;
     cudaError_t e0 = cudaMemsetAsync(tb.flags, 0, sizeof(int), s);
     if (e0 != cudaSuccess) return e0;
-    tc_scale_kernel<<<1, 128, 0, s>>>(D, K, pi, mu, var, tb.sd, tb.kap);
+    tc_scale_kernel<<<128, 128, 0, s>>>(D, K, pi, mu, var, tb.sd, tb.kap);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     tc_prepare_kernel<<<pl.Kpad, 128, 0, s>>>(D, K, pi, mu, var, tb.sd, tb.kap, tb.phi_img, tb.plo_img, tb.tk, tb.ck, tb.illb, cond_limit, tb.flags);
@@ -947,48 +964,47 @@ cudaError_t launch_em_tc(cudaStream_t s, const float* X, int64_t n, int D, int K
     p.phi_img = tb.phi_img; p.plo_img = tb.plo_img; p.tk = tb.tk; p.ck = tb.ck; p.sd = tb.sd; p.kap = tb.kap;
     p.illb = tb.illb; p.flags = tb.flags; p.mu = mu; p.w2 = w2; p.c2 = c2;
     p.partial = tb.partial; p.llpart = tb.llpart; p.status = status;
+    p.xg = static_cast<XSlot*>(tb.xg); p.xl = static_cast<XSlot*>(tb.xl);
 #ifdef FLASHGMM_DEBUG
     p.dbg = g_tc_debug;
     p.dbg_clk = g_tc_clk;
 #endif
     cudaError_t e = cudaFuncSetAttribute(em_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    if (pl.CL > 8) return cudaErrorInvalidValue;
+    // exchange slots carry the tile number as their tag: clear what the previous launch left behind
+    const size_t xbytes = (size_t)Q * 4 * pl.CL * 64 * sizeof(XSlot);
+    e = cudaMemsetAsync(tb.xg, 0, xbytes, s);
+    if (e != cudaSuccess) return e;
+    e = cudaMemsetAsync(tb.xl, 0, xbytes, s);
+    if (e != cudaSuccess) return e;
+    // The CTAs of a group wait for one another, so all of them must be resident at once: a cooperative launch either
+    // guarantees that or fails.
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(Q * pl.CL));
     cfg.blockDim = dim3(NTHREADS);
     cfg.dynamicSmemBytes = SMEM_BYTES;
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = (unsigned)pl.CL;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, em_tc_kernel, p);
 }
 
-// Number of clusters of the plan's size that can be resident at once (1 CTA per SM): the persistent grid size.
+// Number of groups (of ceil(K/128) CTAs, one CTA per SM) that can be resident at once: the persistent grid size.
 cudaError_t tc_max_clusters(int D, int K, int* out) {
     const TcPlan pl = tc_plan(D, K, 148);
     cudaError_t e = cudaFuncSetAttribute(em_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(pl.CL * 148));
-    cfg.blockDim = dim3(NTHREADS);
-    cfg.dynamicSmemBytes = SMEM_BYTES;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = (unsigned)pl.CL;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    int n = 0;
-    e = cudaOccupancyMaxActiveClusters(&n, em_tc_kernel, &cfg);
+    int dev = 0, sms = 0, per_sm = 0;
+    e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
-    *out = n;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, em_tc_kernel, NTHREADS, SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    *out = (sms * per_sm) / pl.CL;
     return cudaSuccess;
 }
 

@@ -12,9 +12,9 @@ constexpr float TC_RSCALE = 4096.f;  // responsibilities are scaled by this powe
 constexpr int TC_PCOLS = 258;        // columns of a partial row: 256 statistics columns + N_k of each softmax group
 
 struct TcPlan {
-    int CL;     // CTAs per cluster = ceil(K / 128)
+    int CL;     // CTAs per group = ceil(K / 128)
     int Kpad;   // CL * 128
-    int Q;      // clusters in the persistent grid
+    int Q;      // groups (of CL CTAs) in the persistent grid
     int n_ks;   // k-steps of 8 dimensions
 };
 
@@ -29,6 +29,8 @@ struct TcBuffers {
     int* flags;
     double* partial;
     double* llpart;
+    void* xg;   // exchange slots of the log-sum-exp, [Q][4][CL][64] x 16 bytes
+    void* xl;   // exchange slots of the lower-bound pass
 };
 
 bool tc_supports(int D, int K);

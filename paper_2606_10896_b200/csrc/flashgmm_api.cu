@@ -28,7 +28,7 @@ inline size_t align256(size_t b) { return (b + 255) & ~(size_t)255; }
 
 struct ScratchLayout {
     size_t w2, c2, partials, logZ2, llpart, result, stats, total;
-    size_t tc_phi, tc_plo, tc_tk, tc_ck, tc_sd, tc_kap, tc_illb, tc_flags, tc_partial, tc_llpart, tc_partial_bytes;
+    size_t tc_phi, tc_plo, tc_tk, tc_ck, tc_sd, tc_kap, tc_illb, tc_flags, tc_xg, tc_xl, tc_partial, tc_llpart, tc_partial_bytes;
     bool tc;
 };
 
@@ -45,7 +45,7 @@ ScratchLayout scratch_layout(int D, int K) {
     L.result = take(sizeof(DevResult));
     L.stats = take(((size_t)K + 2 * KD) * 8);
     L.tc = tc_supports(D, K);
-    L.tc_phi = L.tc_plo = L.tc_tk = L.tc_ck = L.tc_sd = L.tc_kap = L.tc_illb = L.tc_flags = L.tc_partial = L.tc_llpart = 0;
+    L.tc_phi = L.tc_plo = L.tc_tk = L.tc_ck = L.tc_sd = L.tc_kap = L.tc_illb = L.tc_flags = L.tc_xg = L.tc_xl = L.tc_partial = L.tc_llpart = 0;
     L.tc_partial_bytes = 0;
     if (L.tc) {
         const TcPlan pl = tc_plan(D, K, 160);       // an upper bound on the number of clusters
@@ -57,6 +57,8 @@ ScratchLayout scratch_layout(int D, int K) {
         L.tc_kap = take(128 * 4);
         L.tc_illb = take((size_t)pl.Kpad * 4);
         L.tc_flags = take(16);
+        L.tc_xg = take((size_t)pl.Q * 4 * pl.CL * 64 * 16);
+        L.tc_xl = take((size_t)pl.Q * 4 * pl.CL * 64 * 16);
         L.tc_partial_bytes = (size_t)pl.Q * pl.Kpad * TC_PCOLS * 8;
         L.tc_partial = take(L.tc_partial_bytes);
         L.tc_llpart = take((size_t)pl.Q * 16);
@@ -114,6 +116,8 @@ struct gmm_ctx {
         b.kap = reinterpret_cast<float*>(scratch + lay.tc_kap);
         b.illb = reinterpret_cast<float*>(scratch + lay.tc_illb);
         b.flags = reinterpret_cast<int*>(scratch + lay.tc_flags);
+        b.xg = scratch + lay.tc_xg;
+        b.xl = scratch + lay.tc_xl;
         b.partial = reinterpret_cast<double*>(scratch + lay.tc_partial);
         b.llpart = reinterpret_cast<double*>(scratch + lay.tc_llpart);
         return b;

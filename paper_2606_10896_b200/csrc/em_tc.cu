@@ -19,8 +19,8 @@
 // Shared memory: P_lo (64 KB, SW128 K-major), two stages of Y (hi and lo planes, SW128; read K-major by the E-step and
 // MN-major by the M-step), exchange buffers, barriers.
 //
-// Warp roles: warps 0-3 softmax (warp w owns TMEM lanes 32w..32w+31), warps 4-7 load X with coalesced 16-byte loads and
-// build the Y planes, warp 8 issues the MMAs.  Every wait is bounded by a wall-clock limit; on expiry the CTA sets
+// Warp roles: warps 0-7 softmax (two warpgroups, each taking 32 of a tile's 64 points; warp w owns TMEM lanes
+// 32 (w mod 4) ...), warps 8-14 load X with coalesced 16-byte loads and build the Y planes, warp 15 issues the MMAs.  Every wait is bounded by a wall-clock limit; on expiry the CTA sets
 // ST_TIMEOUT, all roles leave their loops, TMEM is freed and the kernel returns.
 #include "internal.cuh"
 #include "em_tc.cuh"
@@ -33,8 +33,9 @@ namespace fg {
 namespace {
 
 constexpr int BN = TC_BN;                 // points per tile
-constexpr int NTHREADS = 416;          // 2 softmax warpgroups (even / odd tiles), 1 transform warpgroup, 1 MMA warp
-constexpr int MMA_WARP = 12;
+constexpr int NTHREADS = 512;          // 8 softmax warps, 7 transform warps, 1 MMA warp (16 warps: 128 registers each)
+constexpr int MMA_WARP = 15;
+constexpr int TR_THREADS = 224;
 constexpr float RSCALE = TC_RSCALE;
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 constexpr float ILL_MARGIN = 40.f;     // log2 units: a logit more than this below the best one is negligible (2^-40)
@@ -63,9 +64,11 @@ enum { B_YFULL0 = 0, B_YFULL1, B_YEMPTY0, B_YEMPTY1, B_LFULL0, B_LFULL1, B_RREAD
 #ifdef FLASHGMM_DEBUG
 #define TIC(var) long long var = clock64()
 #define TOC(var, slot) do { if (p.dbg_clk && blockIdx.x == 0) { long long now_ = clock64(); if ((threadIdx.x & 31) == 0) atomicAdd((unsigned long long*)&p.dbg_clk[slot], (unsigned long long)(now_ - var)); var = now_; } } while (0)
+#define TRACE(ev, tile) do { if (p.dbg_trace && blockIdx.x == 0 && (tile) < 64) p.dbg_trace[(tile) * 16 + (ev)] = clock64(); } while (0)
 #else
 #define TIC(var)
 #define TOC(var, slot)
+#define TRACE(ev, tile)
 #endif
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -182,6 +185,39 @@ __device__ __forceinline__ bool xslot_wait(const XSlot* q, uint32_t tag, float& 
     }
 }
 
+// Bounded poll of the CL slots of one point (stride 64 slots between source CTAs): all outstanding loads are issued
+// together, so one round costs one L2 round trip.
+__device__ __forceinline__ bool xslot_wait_all(const XSlot* q, int CL, uint32_t tag, float2 (&e)[8], volatile int* abort_flag,
+                                               int* status) {
+    uint32_t pending = (CL >= 32) ? 0xffffffffu : ((1u << CL) - 1u);
+#pragma unroll
+    for (int c = 0; c < 8; ++c) e[c] = make_float2(-CUDART_INF_F, 0.f);
+    unsigned long long t0 = 0;
+    for (int it = 0;; ++it) {
+        uint32_t v[8][4];
+#pragma unroll
+        for (int c = 0; c < 8; ++c)
+            if (pending & (1u << c)) xslot_load(q + c * 64, v[c]);
+#pragma unroll
+        for (int c = 0; c < 8; ++c)
+            if ((pending & (1u << c)) && v[c][1] == tag && v[c][3] == tag) {
+                e[c] = make_float2(__uint_as_float(v[c][0]), __uint_as_float(v[c][2]));
+                pending &= ~(1u << c);
+            }
+        if (pending == 0u) return true;
+        if (*abort_flag) return false;
+        if ((it & 15) == 15) {
+            const unsigned long long now = gtime();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > WAIT_LIMIT_NS) {
+                *abort_flag = 1;
+                atomicOr(status, ST_TIMEOUT);
+                return false;
+            }
+        }
+    }
+}
+
 __device__ __forceinline__ void named_bar_sync(int id, int count) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
 }
@@ -205,6 +241,13 @@ __device__ __forceinline__ void tmem_st32(uint32_t addr, const uint32_t (&v)[32]
           "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]), "r"(v[16]), "r"(v[17]),
           "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]), "r"(v[24]), "r"(v[25]), "r"(v[26]),
           "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t addr, const uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+        ::"r"(addr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]),
+          "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
         : "memory");
 }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
@@ -232,6 +275,18 @@ __device__ __forceinline__ void warp_reduce_scatter(const float (&v)[64], float 
     bfly_round<2, IS_MAX>(d, out, lane & 1, 1);
 }
 
+// 32-value variant: afterwards lane l holds the reduction for point l.
+template <bool IS_MAX>
+__device__ __forceinline__ void warp_reduce_scatter32(const float (&v)[32], float& out, int lane) {
+    float a[16], b[8], c[4], d[2], e[1];
+    bfly_round<16, IS_MAX>(v, a, lane & 16, 16);
+    bfly_round<8, IS_MAX>(a, b, lane & 8, 8);
+    bfly_round<4, IS_MAX>(b, c, lane & 4, 4);
+    bfly_round<2, IS_MAX>(c, d, lane & 2, 2);
+    bfly_round<1, IS_MAX>(d, e, lane & 1, 1);
+    out = e[0];
+}
+
 __device__ __forceinline__ uint32_t pack_h2(__half lo, __half hi) {
     return (uint32_t)__half_as_ushort(lo) | ((uint32_t)__half_as_ushort(hi) << 16);
 }
@@ -239,7 +294,7 @@ __device__ __forceinline__ uint32_t pack_h2(__half lo, __half hi) {
 struct TcKernelParams {
     const float* X;
     int64_t n;
-    int D, K, CL, Q, n_ks, flush;
+    int D, K, CL, Q, n_ks, flush, order;
     const uint32_t* phi_img;       // [CL][128 lanes][128] packed fp16 pairs
     const unsigned char* plo_img;  // [CL][65536] shared-memory image (SW128, K-major)
     const float* tk;               // [CL*128]
@@ -259,6 +314,7 @@ struct TcKernelParams {
 #ifdef FLASHGMM_DEBUG
     float* dbg;      // [Kpad][64] log2 z of the first tile
     long long* dbg_clk;   // per-phase cycle counters of CTA 0
+    long long* dbg_trace; // [64 tiles][16 events] clock64 stamps of CTA 0
 #endif
 };
 
@@ -285,10 +341,10 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
         abort_s = 0;
         decision_s[0] = 0;
         decision_s[1] = 0;
-        bar_init(BAR(B_YFULL0), 128);  bar_init(BAR(B_YFULL1), 128);
+        bar_init(BAR(B_YFULL0), TR_THREADS);  bar_init(BAR(B_YFULL1), TR_THREADS);
         bar_init(BAR(B_YEMPTY0), 1);   bar_init(BAR(B_YEMPTY1), 1);
         bar_init(BAR(B_LFULL0), 1);    bar_init(BAR(B_LFULL1), 1);
-        bar_init(BAR(B_RREADY0), 128); bar_init(BAR(B_RREADY1), 128);
+        bar_init(BAR(B_RREADY0), 256); bar_init(BAR(B_RREADY1), 256);
         bar_init(BAR(B_ACCFULL), 1);   bar_init(BAR(B_ACCFREE), 128);
         bar_init(BAR(B_FINAL), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -333,23 +389,25 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
 
     if (warp < 8) {
         // =========================== softmax warps ===========================
-        // Two warpgroups: group g (warps 4g..4g+3) handles the local tiles with i % 2 == g, i.e. always stage / logits
-        // buffer g, so a tile's softmax has two tile periods of the tensor pipe to finish.
+        // Two warpgroups share every tile: group g (warps 4g..4g+3) takes points 32g..32g+31, so the latency between the
+        // E-step and the M-step of a tile is that of a 32-point softmax (latency, not throughput, is what the tensor
+        // pipe waits for).
         const int grp = warp >> 2, wq = warp & 3, gtid = tid & 127;
+        const int p0 = 32 * grp;                                // first point of this group within the tile
         const uint32_t lane_addr = ((uint32_t)(wq * 32)) << 16;
         const int kloc = gtid;                                  // component within the slice
         const float tk = p.tk[rank * 128 + kloc];
         const float ck = p.ck[rank * 128 + kloc];
         const float illb = p.illb[rank * 128 + kloc];
         const bool any_ill = p.flags[0] != 0;
-        float* gather = reinterpret_cast<float*>(smem + SM_GATHER) + warp * 64;
-        float2* ws = reinterpret_cast<float2*>(smem + SM_WS) + grp * 256;      // [4][64] per group
-        float* fac = reinterpret_cast<float*>(smem + SM_FAC) + grp * 256;      // [4][64] per group
+        float* gather = reinterpret_cast<float*>(smem + SM_GATHER) + warp * 32;    // [8 warps][32]
+        float2* ws = reinterpret_cast<float2*>(smem + SM_WS) + grp * 128;          // [4][32] per group
+        float* fac = reinterpret_cast<float*>(smem + SM_FAC) + grp * 128;          // [4][32] per group
         XSlot* xg = p.xg + (size_t)cluster_id * 4 * p.CL * 64;             // [4][CL][64] ring of exchange slots
         XSlot* xl = p.xl + (size_t)cluster_id * 4 * p.CL * 64;             // same, for the lower-bound exchange
         float nk_acc = 0.f;
         double ll_acc = 0.0;
-        // partial layout [cluster][column][component]: the 32 lanes of a warp touch 32 consecutive doubles; every address
+        // partial layout [group][column][component]: the 32 lanes of a warp touch 32 consecutive doubles; every address
         // belongs to exactly one thread of the grid, so the reductions below are deterministic
         const size_t pstride = (size_t)p.CL * 128;
         double* prow = p.partial + (size_t)cluster_id * TC_PCOLS * pstride + rank * 128 + kloc;
@@ -357,91 +415,81 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
 
         // Softmax threads leave the loop only at the uniform decision point after named barrier 2: a thread that
         // left earlier would strand the others in a hardware barrier.
-        for (int64_t i = grp; i < ntl; i += 2) {
-            const int s = grp;
+        for (int64_t i = 0; i < ntl; ++i) {
+            const int s = (int)(i & 1);
             const uint32_t ph = (uint32_t)((i >> 1) & 1);
             const int64_t tile = cluster_id + i * p.Q;
             const int64_t row0 = tile * BN;
-            const int nvalid = (int)((p.n - row0 < BN) ? (p.n - row0) : BN);
+            const int nvalid = (int)((p.n - row0 < BN) ? (p.n - row0) : BN) - p0;     // valid points of this group's half
 
             TIC(tk_);
             if (!bar_wait(BAR(B_LFULL0 + s), ph, abort_flag, p.status, false)) alive = false;
             TOC(tk_, 0);
+            if (gtid == 0) TRACE(0, i);
             fence_after();
-            float l[64];
+            float l[32];
             {
-                uint32_t v0[32], v1[32];
-                tmem_ld32(T_LOG + s * 64 + lane_addr, v0);
-                tmem_ld32(T_LOG + s * 64 + lane_addr + 32, v1);
+                uint32_t v0[32];
+                tmem_ld32(T_LOG + s * 64 + p0 + lane_addr, v0);
                 tmem_wait_ld();
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    l[j] = fmaf(__uint_as_float(v0[j]), tk, ck);
-                    l[32 + j] = fmaf(__uint_as_float(v1[j]), tk, ck);
-                }
+                for (int j = 0; j < 32; ++j) l[j] = fmaf(__uint_as_float(v0[j]), tk, ck);
             }
 #ifdef FLASHGMM_DEBUG
             if (p.dbg && cluster_id == 0 && i == 0)
-                for (int j = 0; j < 64; ++j) p.dbg[(size_t)(rank * 128 + kloc) * 64 + j] = l[j];
+                for (int j = 0; j < 32; ++j) p.dbg[(size_t)(rank * 128 + kloc) * 64 + p0 + j] = l[j];
 #endif
             TOC(tk_, 16);
-            float red[2];
-            // Ill-conditioned components (sum_d mu^2 / var too large for the 22-bit expanded form, e.g. a component
-            // that collapsed onto a few points): wherever such a component is within reach of the warp's maximum for a
-            // point, its logit is recomputed exactly with direct differences in fp32, the whole warp working on one
-            // (component, point) pair at a time.  Rare by construction: a tight component is competitive for few points.
+            float red;
             // Ill-conditioned components (sum_d mu^2 / var too large for the 22-bit expanded form, e.g. a component
             // collapsed onto a few points): their approximate logits carry an error of up to E_k.  A (component, point)
             // pair can only matter if its upper bound l + E_k reaches the best LOWER bound max_k' (l - E_k') over ALL K
-            // components minus the 2^-40 margin, so the lower bounds are maximised over the cluster first (one extra
+            // components minus the 2^-40 margin, so the lower bounds are maximised over the group first (one extra
             // exchange, only in launches that have such components).  Pairs that pass are recomputed exactly with
             // direct differences in fp32, the whole warp working on one pair at a time; the rest are provably negligible.
             if (any_ill) {
-                float* lbw = reinterpret_cast<float*>(smem + SM_LBW) + grp * 256;       // [4][64]
-                float* lbg = reinterpret_cast<float*>(smem + SM_LBG) + grp * 64;        // [64]
+                float* lbw = reinterpret_cast<float*>(smem + SM_LBW) + grp * 128;       // [4][32]
+                float* lbg = reinterpret_cast<float*>(smem + SM_LBG) + grp * 32;        // [32]
                 if (illb > 0.f) {
 #pragma unroll
-                    for (int j = 0; j < 64; ++j) l[j] -= illb;
+                    for (int j = 0; j < 32; ++j) l[j] -= illb;
                 }
-                warp_reduce_scatter<true>(l, red, lane);
+                warp_reduce_scatter32<true>(l, red, lane);
                 if (illb > 0.f) {
 #pragma unroll
-                    for (int j = 0; j < 64; ++j) l[j] += illb;      // (restores l up to ulp(E_k): irrelevant next to E_k)
+                    for (int j = 0; j < 32; ++j) l[j] += illb;      // (restores l up to ulp(E_k): irrelevant next to E_k)
                 }
-                reinterpret_cast<float2*>(lbw + wq * 64)[lane] = make_float2(red[0], red[1]);
+                lbw[wq * 32 + lane] = red;
                 named_bar_sync(7 + 2 * grp, 128);
-                if (gtid < 64) {
-                    const float m4 = fmaxf(fmaxf(lbw[gtid], lbw[64 + gtid]), fmaxf(lbw[128 + gtid], lbw[192 + gtid]));
+                if (gtid < 32) {
+                    const float m4 = fmaxf(fmaxf(lbw[gtid], lbw[32 + gtid]), fmaxf(lbw[64 + gtid], lbw[96 + gtid]));
                     const uint32_t tag = (uint32_t)(i + 1);
-                    XSlot* ring = xl + (size_t)(i & 3) * p.CL * 64;
-                    xslot_write(ring + rank * 64 + gtid, m4, 0.f, tag);
+                    XSlot* ring = xl + (size_t)(i & 3) * p.CL * 64 + p0 + gtid;
+                    xslot_write(ring + rank * 64, m4, 0.f, tag);
+                    float2 e[8];
+                    if (!xslot_wait_all(ring, p.CL, tag, e, abort_flag, p.status)) alive = false;
                     float mg = -CUDART_INF_F;
-                    for (int c = 0; c < p.CL; ++c) {
-                        float a = -CUDART_INF_F, b = 0.f;
-                        if (!xslot_wait(ring + c * 64 + gtid, tag, a, b, abort_flag, p.status)) alive = false;
-                        mg = fmaxf(mg, a);
-                    }
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) mg = fmaxf(mg, e[c].x);
                     lbg[gtid] = mg;
                 }
                 named_bar_sync(8 + 2 * grp, 128);
                 if (__any_sync(0xffffffffu, illb > 0.f)) {
                     const int kglob = (int)rank * 128 + kloc;
-                    uint32_t mlo = 0, mhi = 0;
+                    uint32_t mlo = 0;
                     if (illb > 0.f) {
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) {
+                        for (int j = 0; j < 32; ++j)
                             if (j < nvalid && l[j] + illb >= lbg[j] - ILL_MARGIN) mlo |= 1u << j;
-                            if (32 + j < nvalid && l[32 + j] + illb >= lbg[32 + j] - ILL_MARGIN) mhi |= 1u << j;
-                        }
                     }
                     for (;;) {
-                        const uint32_t ballot = __ballot_sync(0xffffffffu, (mlo | mhi) != 0u);
+                        const uint32_t ballot = __ballot_sync(0xffffffffu, mlo != 0u);
                         if (ballot == 0u) break;
                         const int src = __ffs(ballot) - 1;
-                        int j = mlo ? (__ffs(mlo) - 1) : (32 + __ffs(mhi) - 1);
+                        int j = __ffs(mlo) - 1;
                         j = __shfl_sync(0xffffffffu, j, src);
                         const int kk = __shfl_sync(0xffffffffu, kglob, src);
-                        const float* xr = p.X + (row0 + j) * p.D;
+                        const float* xr = p.X + (row0 + p0 + j) * p.D;
                         const float* mr = p.mu + (size_t)kk * p.D;
                         const float* wr = p.w2 + (size_t)kk * p.D;
                         float q = 0.f;
@@ -454,21 +502,20 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                         const float val = __ldg(p.c2 + kk) - q;
                         if (lane == src) {
 #pragma unroll
-                            for (int jj = 0; jj < 64; ++jj)
+                            for (int jj = 0; jj < 32; ++jj)
                                 if (jj == j) l[jj] = val;
-                            if (j < 32) mlo &= ~(1u << j); else mhi &= ~(1u << (j - 32));
+                            mlo &= ~(1u << j);
                         }
                     }
                 }
             }
-            // warp-level max per point, all-gathered through shared memory
-            warp_reduce_scatter<true>(l, red, lane);
-            reinterpret_cast<float2*>(gather)[lane] = make_float2(red[0], red[1]);
+            // warp-level max per point (lane j ends up with point j), all-gathered through shared memory
+            warp_reduce_scatter32<true>(l, red, lane);
+            gather[lane] = red;
             __syncwarp();
             TOC(tk_, 17);
-            const float mw_mine0 = red[0], mw_mine1 = red[1];
 #pragma unroll
-            for (int j = 0; j < 64; j += 4) {
+            for (int j = 0; j < 32; j += 4) {
                 const float4 m4 = *reinterpret_cast<const float4*>(gather + j);
                 const float m0 = (m4.x == -CUDART_INF_F) ? 0.f : m4.x;
                 const float m1 = (m4.y == -CUDART_INF_F) ? 0.f : m4.y;
@@ -481,17 +528,18 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
             }
             __syncwarp();
             TOC(tk_, 18);
-            float sred[2];
-            warp_reduce_scatter<false>(l, sred, lane);
-            *reinterpret_cast<float4*>(&ws[wq * 64 + 2 * lane]) = make_float4(mw_mine0, sred[0], mw_mine1, sred[1]);
+            float sred;
+            warp_reduce_scatter32<false>(l, sred, lane);
+            ws[wq * 32 + lane] = make_float2(red, sred);
             TOC(tk_, 1);
             named_bar_sync(1 + 2 * grp, 128);
             TOC(tk_, 2);
-            if (gtid < 64) {
+            if (gtid == 0) TRACE(1, i);
+            if (gtid < 32) {
                 const int pt = gtid;
                 float2 w4[4];
 #pragma unroll
-                for (int w = 0; w < 4; ++w) w4[w] = ws[w * 64 + pt];
+                for (int w = 0; w < 4; ++w) w4[w] = ws[w * 32 + pt];
                 float mc = fmaxf(fmaxf(w4[0].x, w4[1].x), fmaxf(w4[2].x, w4[3].x));
                 const float mc_safe = (mc == -CUDART_INF_F) ? 0.f : mc;
                 float sc = 0.f;
@@ -500,20 +548,16 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                     sc += (w4[w].x == -CUDART_INF_F) ? 0.f : w4[w].y * fast_ex2(w4[w].x - mc_safe);
                 // publish (m, s) of this CTA's 128 components, then collect the group's
                 const uint32_t tag = (uint32_t)(i + 1);
-                XSlot* ring = xg + (size_t)(i & 3) * p.CL * 64;
-                xslot_write(ring + rank * 64 + pt, mc, sc, tag);
+                XSlot* ring = xg + (size_t)(i & 3) * p.CL * 64 + p0 + pt;
+                xslot_write(ring + rank * 64, mc, sc, tag);
                 TOC(tk_, 3);
-                float mi = -CUDART_INF_F;
                 float2 e[8];
+                if (!xslot_wait_all(ring, p.CL, tag, e, abort_flag, p.status)) alive = false;
+                float mi = -CUDART_INF_F;
 #pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    e[c] = make_float2(-CUDART_INF_F, 0.f);
-                    if (c < p.CL) {
-                        if (!xslot_wait(ring + c * 64 + pt, tag, e[c].x, e[c].y, abort_flag, p.status)) alive = false;
-                    }
-                    mi = fmaxf(mi, e[c].x);
-                }
+                for (int c = 0; c < 8; ++c) mi = fmaxf(mi, e[c].x);
                 TOC(tk_, 4);
+                if (gtid == 0) TRACE(2, i);
                 const float mi_safe = (mi == -CUDART_INF_F) ? 0.f : mi;
                 float Z = 0.f;
 #pragma unroll
@@ -523,21 +567,22 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                 const float inv = (valid && Z > 0.f) ? (RSCALE / Z) : 0.f;
 #pragma unroll
                 for (int w = 0; w < 4; ++w)
-                    fac[w * 64 + pt] = (w4[w].x == -CUDART_INF_F) ? 0.f : fast_ex2(w4[w].x - mi_safe) * inv;
+                    fac[w * 32 + pt] = (w4[w].x == -CUDART_INF_F) ? 0.f : fast_ex2(w4[w].x - mi_safe) * inv;
                 if (rank == 0 && valid) ll_acc += (double)(mi + log2f(Z));
             }
             if (gtid == 0) decision_s[grp] = *abort_flag;
             TOC(tk_, 5);
             named_bar_sync(2 + 2 * grp, 128);
             TOC(tk_, 6);
+            if (gtid == 0) TRACE(3, i);
             if (decision_s[grp]) break;
             // responsibilities: r = p * fac, split into fp16 hi + lo, written over the logits as the M-step A operand
             {
-                uint32_t hi[32], lo[32];
-                const float* fw = fac + wq * 64;
+                uint32_t hi[16], lo[16];
+                const float* fw = fac + wq * 32;
                 float nsum = 0.f;
 #pragma unroll
-                for (int j = 0; j < 64; j += 4) {
+                for (int j = 0; j < 32; j += 4) {
                     const float4 f4 = *reinterpret_cast<const float4*>(fw + j);
                     const float r0 = l[j] * f4.x, r1 = l[j + 1] * f4.y, r2 = l[j + 2] * f4.z, r3 = l[j + 3] * f4.w;
                     const __half2 h01 = __floats2half2_rn(r0, r1), h23 = __floats2half2_rn(r2, r3);
@@ -551,19 +596,21 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                     lo[j / 2 + 1] = *reinterpret_cast<const uint32_t*>(&g23);
                 }
                 nk_acc += nsum;
-                tmem_st32(T_LOG + s * 64 + lane_addr, hi);
-                tmem_st32(T_LOG + s * 64 + lane_addr + 32, lo);
+                // each group overwrites only the 32 columns its own logits came from: [r_hi (16) | r_lo (16)]
+                tmem_st16(T_LOG + s * 64 + p0 + lane_addr, hi);
+                tmem_st16(T_LOG + s * 64 + p0 + 16 + lane_addr, lo);
                 tmem_wait_st();
             }
             fence_before();
             bar_arrive(BAR(B_RREADY0 + s));
             TOC(tk_, 7);
+            if (gtid == 0) TRACE(4, i);
 
-            // periodic flush of the TMEM accumulators into float64 partials: by the group that owns the last tile of the
-            // pair; the flush index (hence the barrier parity) follows from the tile index alone
+            // periodic flush of the TMEM accumulators into float64 partials, by group 1, after the second tile of a pair
+            // (or the last tile); the flush index (hence the barrier parity) follows from the tile index alone
             const bool pair_end = (i & 1) || (i + 1 == ntl);
             const int64_t pair_next = (i | 1) + 1;
-            if (pair_end && ((pair_next % p.flush) == 0 || pair_next >= ntl)) {
+            if (grp == 1 && pair_end && ((pair_next % p.flush) == 0 || pair_next >= ntl)) {
                 const uint32_t fpar = (uint32_t)(((pair_next - 1) / p.flush) & 1);
                 if (!bar_wait(BAR(B_ACCFULL), fpar, abort_flag, p.status, false)) alive = false;
                 fence_after();
@@ -579,65 +626,61 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                 bar_arrive(BAR(B_ACCFREE));
                 TOC(tk_, 8);
             }
-            // N_k of this group's tiles has its own column, flushed on the group's own cadence
-            if ((((i >> 1) + 1) % 32) == 0 || i + 2 >= ntl) {
+            // N_k of this group's points has its own column
+            if (((i + 1) % 64) == 0 || i + 1 >= ntl) {
                 atomicAdd(prow + (size_t)(256 + grp) * pstride, (double)nk_acc);
                 nk_acc = 0.f;
             }
         }
         if (rank == 0) {
-            double* lls = reinterpret_cast<double*>(smem + SM_LL) + grp * 64;
-            if (gtid < 64) lls[gtid] = ll_acc;
+            double* lls = reinterpret_cast<double*>(smem + SM_LL) + grp * 32;
+            if (gtid < 32) lls[gtid] = ll_acc;
             named_bar_sync(5 + grp, 128);
             if (gtid == 0) {
                 double sum = 0.0;
-                for (int j = 0; j < 64; ++j) sum += lls[j];
+                for (int j = 0; j < 32; ++j) sum += lls[j];
                 p.llpart[cluster_id * 2 + grp] = sum * 0.69314718055994530942;
             }
         }
     } else if (warp < MMA_WARP) {
         // =========================== transform warps: X -> Y planes ===========================
+        // 224 threads share the 1024 (point, 8-dimension group) units of a tile: unit u = tau + 224 n, point u / 16,
+        // group u % 16 (16 consecutive threads read one row: coalesced 32-byte pieces).  A tile is loaded and converted
+        // into its four fp16 planes in registers BEFORE the wait for the stage, so that only the shared-memory stores
+        // sit between the release of a stage and its next use.
         const int tau = tid - 256;
-        const int pt = tau >> 1, half = tau & 1;
         const bool vec_ok = (p.D % 4 == 0) && ((reinterpret_cast<uintptr_t>(p.X) & 15) == 0);
+        constexpr int NU = 5;                               // ceil(1024 / 224)
         for (int64_t i = 0; i < ntl; ++i) {
             const int s = (int)(i & 1);
             const uint32_t ph = (uint32_t)((i >> 1) & 1);
-            const int64_t row = (cluster_id + i * p.Q) * BN + pt;
-            const bool row_ok = row < p.n;
-            const float* xr = p.X + row * p.D;
+            const int64_t row_base = (cluster_id + i * p.Q) * BN;
             unsigned char* yhi = smem + SM_Y + s * SM_YSTAGE;
             unsigned char* ylo = yhi + SM_YLO;
-            float4 xa[8], xb[8];
-            const bool fast = row_ok && vec_ok && (half * 64 + 64 <= p.D);
-            if (fast) {
+            float4 xa[NU], xb[NU];
 #pragma unroll
-                for (int g = 0; g < 8; ++g) {
-                    xa[g] = __ldg(reinterpret_cast<const float4*>(xr + half * 64 + g * 8));
-                    xb[g] = __ldg(reinterpret_cast<const float4*>(xr + half * 64 + g * 8 + 4));
-                }
-            } else {
-#pragma unroll
-                for (int g = 0; g < 8; ++g) {
-                    const int d0 = half * 64 + g * 8;
+            for (int n = 0; n < NU; ++n) {
+                const int u = tau + n * TR_THREADS;
+                const int pt = u >> 4, ks = u & 15, d0 = ks * 8;
+                const int64_t row = row_base + pt;
+                const bool row_ok = (u < 1024) && (row < p.n);
+                const float* xr = p.X + row * p.D;
+                if (row_ok && vec_ok && d0 + 8 <= p.D) {
+                    xa[n] = __ldg(reinterpret_cast<const float4*>(xr + d0));
+                    xb[n] = __ldg(reinterpret_cast<const float4*>(xr + d0 + 4));
+                } else {
                     float x[8];
 #pragma unroll
                     for (int j = 0; j < 8; ++j) x[j] = (row_ok && d0 + j < p.D) ? __ldg(xr + d0 + j) : 0.f;
-                    xa[g] = make_float4(x[0], x[1], x[2], x[3]);
-                    xb[g] = make_float4(x[4], x[5], x[6], x[7]);
+                    xa[n] = make_float4(x[0], x[1], x[2], x[3]);
+                    xb[n] = make_float4(x[4], x[5], x[6], x[7]);
                 }
             }
-            // the loads above are in flight while this thread waits for the stage to be released
-            TIC(tt_);
-            if (i >= 2) {
-                if (!bar_wait(BAR(B_YEMPTY0 + s), ph ^ 1, abort_flag, p.status, false)) break;
-            }
-            TOC(tt_, 10);
+            uint4 vxh[NU], vxl[NU], vqh[NU], vql[NU];
 #pragma unroll
-            for (int g = 0; g < 8; ++g) {
-                const int ks = half * 8 + g;
-                const int d0 = ks * 8;
-                const float x[8] = {xa[g].x, xa[g].y, xa[g].z, xa[g].w, xb[g].x, xb[g].y, xb[g].z, xb[g].w};
+            for (int n = 0; n < NU; ++n) {
+                const int d0 = ((tau + n * TR_THREADS) & 15) * 8;
+                const float x[8] = {xa[n].x, xa[n].y, xa[n].z, xa[n].w, xb[n].x, xb[n].y, xb[n].z, xb[n].w};
                 uint32_t xh[4], xl[4], qh[4], ql[4];
 #pragma unroll
                 for (int j = 0; j < 8; j += 2) {
@@ -656,19 +699,37 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                     qh[j / 2] = *reinterpret_cast<const uint32_t*>(&sq);
                     ql[j / 2] = *reinterpret_cast<const uint32_t*>(&t2);
                 }
-                // 16-byte chunk index in the point's 512-byte row: 2 ks (x) and 2 ks + 1 (x^2)
-                const int atom = ks >> 2;
-                const int cx = ((2 * (ks & 3)) ^ (pt & 7)) << 4;
-                const int cq = ((2 * (ks & 3) + 1) ^ (pt & 7)) << 4;
-                const int base = atom * 8192 + pt * 128;
-                *reinterpret_cast<uint4*>(yhi + base + cx) = make_uint4(xh[0], xh[1], xh[2], xh[3]);
-                *reinterpret_cast<uint4*>(yhi + base + cq) = make_uint4(qh[0], qh[1], qh[2], qh[3]);
-                *reinterpret_cast<uint4*>(ylo + base + cx) = make_uint4(xl[0], xl[1], xl[2], xl[3]);
-                *reinterpret_cast<uint4*>(ylo + base + cq) = make_uint4(ql[0], ql[1], ql[2], ql[3]);
+                vxh[n] = make_uint4(xh[0], xh[1], xh[2], xh[3]);
+                vxl[n] = make_uint4(xl[0], xl[1], xl[2], xl[3]);
+                vqh[n] = make_uint4(qh[0], qh[1], qh[2], qh[3]);
+                vql[n] = make_uint4(ql[0], ql[1], ql[2], ql[3]);
+            }
+            TIC(tt_);
+            if (i >= 2) {
+                if (!bar_wait(BAR(B_YEMPTY0 + s), ph ^ 1, abort_flag, p.status, false)) break;
+            }
+            TOC(tt_, 10);
+            if (tau == 0) TRACE(5, i);
+#pragma unroll
+            for (int n = 0; n < NU; ++n) {
+                const int u = tau + n * TR_THREADS;
+                if (u < 1024) {
+                    const int pt = u >> 4, ks = u & 15;
+                    // 16-byte chunk index in the point's 512-byte row: 2 ks (x) and 2 ks + 1 (x^2)
+                    const int atom = ks >> 2;
+                    const int cx = ((2 * (ks & 3)) ^ (pt & 7)) << 4;
+                    const int cq = ((2 * (ks & 3) + 1) ^ (pt & 7)) << 4;
+                    const int base = atom * 8192 + pt * 128;
+                    *reinterpret_cast<uint4*>(yhi + base + cx) = vxh[n];
+                    *reinterpret_cast<uint4*>(yhi + base + cq) = vqh[n];
+                    *reinterpret_cast<uint4*>(ylo + base + cx) = vxl[n];
+                    *reinterpret_cast<uint4*>(ylo + base + cq) = vql[n];
+                }
             }
             fence_async_smem();
             bar_arrive(BAR(B_YFULL0 + s));
             TOC(tt_, 11);
+            if (tau == 0) TRACE(6, i);
         }
     } else if (lane == 0) {
         // =========================== MMA issuer (one thread) ===========================
@@ -684,6 +745,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
             TIC(tm_);
             if (!bar_wait(BAR(B_YFULL0 + s), ph, abort_flag, p.status, false)) return false;
             TOC(tm_, 12);
+            TRACE(7, i);
             fence_after();
             const uint32_t yhi = smem_u32(smem + SM_Y + s * SM_YSTAGE), ylo = yhi + SM_YLO;
             const uint32_t d = T_LOG + s * 64;
@@ -698,6 +760,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                 mma_ts(d, T_PHI + ks * 8, make_desc(yhi + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024), id_e, 1);
             mma_commit(BAR(B_LFULL0 + s));
             TOC(tm_, 13);
+            TRACE(8, i);
             return true;
         };
         auto issue_M = [&](int64_t i) -> bool {
@@ -706,35 +769,59 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
             TIC(tm_);
             if (!bar_wait(BAR(B_RREADY0 + s), ph, abort_flag, p.status, false)) return false;
             TOC(tm_, 14);
+            TRACE(9, i);
             fence_after();
             const uint32_t yhi = smem_u32(smem + SM_Y + s * SM_YSTAGE), ylo = yhi + SM_YLO;
-            const uint32_t rhi = T_LOG + s * 64, rlo = rhi + 32;
+            // A operand layout in the logits buffer: points 0-31 -> columns [0,16) r_hi, [16,32) r_lo; points 32-63 -> +32
+            const uint32_t rbase = T_LOG + s * 64;
+            auto r_hi = [&](int ks) { return rbase + (ks >> 1) * 32 + (ks & 1) * 8; };
             for (int ks = 0; ks < BN / 16; ++ks) {
-                mma_ts(T_ACC, rhi + ks * 8, make_desc(yhi + ks * 2048, 8192, 1024), id_m, acc_valid || ks > 0);
+                mma_ts(T_ACC, r_hi(ks), make_desc(yhi + ks * 2048, 8192, 1024), id_m, acc_valid || ks > 0);
             }
             acc_valid = true;
-            for (int ks = 0; ks < BN / 16; ++ks) mma_ts(T_ACC, rhi + ks * 8, make_desc(ylo + ks * 2048, 8192, 1024), id_m, 1);
-            for (int ks = 0; ks < BN / 16; ++ks) mma_ts(T_ACC, rlo + ks * 8, make_desc(yhi + ks * 2048, 8192, 1024), id_m, 1);
+            for (int ks = 0; ks < BN / 16; ++ks) mma_ts(T_ACC, r_hi(ks), make_desc(ylo + ks * 2048, 8192, 1024), id_m, 1);
+            for (int ks = 0; ks < BN / 16; ++ks) mma_ts(T_ACC, r_hi(ks) + 16, make_desc(yhi + ks * 2048, 8192, 1024), id_m, 1);
             mma_commit(BAR(B_YEMPTY0 + s));
             TOC(tm_, 15);
+            TRACE(10, i);
             return true;
         };
-        // Issue order per pair of tiles: E(a) E(b) M(a) M(b).  (The interleaved order M(i) E(i+2) M(i+1) ... was measured
-        // slower: it puts the Y-stage refill between every M and the following E on the tensor pipe's critical path.)
-        for (int64_t i = 0; i < ntl && alive; i += 2) {
-            const bool has2 = i + 1 < ntl;
-            alive = issue_E(i);
-            if (alive && has2) alive = issue_E(i + 1);
-            if (alive) alive = issue_M(i);
-            if (alive && has2) alive = issue_M(i + 1);
-            if (!alive) break;
-            const int64_t pair_next = i + 2;
-            if ((pair_next % p.flush) == 0 || pair_next >= ntl) {
-                mma_commit(BAR(B_ACCFULL));
-                if (!bar_wait(BAR(B_ACCFREE), accfree_parity, abort_flag, p.status, false)) { alive = false; break; }
-                accfree_parity ^= 1;
-                fence_after();
-                acc_valid = false;
+        if (p.order == 0) {
+            // Issue order per pair of tiles: E(a) E(b) M(a) M(b).
+            for (int64_t i = 0; i < ntl && alive; i += 2) {
+                const bool has2 = i + 1 < ntl;
+                alive = issue_E(i);
+                if (alive && has2) alive = issue_E(i + 1);
+                if (alive) alive = issue_M(i);
+                if (alive && has2) alive = issue_M(i + 1);
+                if (!alive) break;
+                const int64_t pair_next = i + 2;
+                if ((pair_next % p.flush) == 0 || pair_next >= ntl) {
+                    mma_commit(BAR(B_ACCFULL));
+                    if (!bar_wait(BAR(B_ACCFREE), accfree_parity, abort_flag, p.status, false)) { alive = false; break; }
+                    accfree_parity ^= 1;
+                    fence_after();
+                    acc_valid = false;
+                }
+            }
+        } else {
+            // Interleaved order E(0) E(1) | M(0) E(2) | M(1) E(3) | ...: M(i) must precede E(i+2) (two logits buffers, two
+            // Y stages); the softmax of tile i+1 overlaps E(i+2).
+            if (ntl > 0) alive = issue_E(0);
+            if (alive && ntl > 1) alive = issue_E(1);
+            for (int64_t i = 0; i < ntl && alive; ++i) {
+                alive = issue_M(i);
+                if (!alive) break;
+                const bool pair_end = (i & 1) || (i + 1 == ntl);
+                const int64_t pair_next = (i | 1) + 1;
+                if (pair_end && ((pair_next % p.flush) == 0 || pair_next >= ntl)) {
+                    mma_commit(BAR(B_ACCFULL));
+                    if (!bar_wait(BAR(B_ACCFREE), accfree_parity, abort_flag, p.status, false)) { alive = false; break; }
+                    accfree_parity ^= 1;
+                    fence_after();
+                    acc_valid = false;
+                }
+                if (i + 2 < ntl) alive = issue_E(i + 2);
             }
         }
         // drain: every MMA issued by this thread has completed before TMEM is released
@@ -913,9 +1000,14 @@ __global__ void tc_reduce_kernel(int D, int K, int Kpad, int Q, const double* __
 #ifdef FLASHGMM_DEBUG
 float* g_tc_debug = nullptr;
 long long* g_tc_clk = nullptr;
+long long* g_tc_trace = nullptr;
+extern "C" void gmm_debug_set_trace(long long* p) { g_tc_trace = p; }
 extern "C" void gmm_debug_set_buffer(float* p) { g_tc_debug = p; }
 extern "C" void gmm_debug_set_clk(long long* p) { g_tc_clk = p; }
 #endif
+
+int g_tc_order = 1;
+void tc_set_order(int o) { g_tc_order = o; }
 
 bool tc_supports(int D, int K) { return D >= 1 && D <= 128 && K >= 1 && K <= 1024; }
 
@@ -961,6 +1053,7 @@ cudaError_t launch_em_tc(cudaStream_t s, const float* X, int64_t n, int D, int K
     TcKernelParams p;
     p.X = X; p.n = n; p.D = D; p.K = K; p.CL = pl.CL; p.Q = Q; p.n_ks = pl.n_ks;
     p.flush = (flush_tiles < 2) ? 2 : (flush_tiles & ~1);
+    p.order = g_tc_order;
     p.phi_img = tb.phi_img; p.plo_img = tb.plo_img; p.tk = tb.tk; p.ck = tb.ck; p.sd = tb.sd; p.kap = tb.kap;
     p.illb = tb.illb; p.flags = tb.flags; p.mu = mu; p.w2 = w2; p.c2 = c2;
     p.partial = tb.partial; p.llpart = tb.llpart; p.status = status;
@@ -968,6 +1061,7 @@ cudaError_t launch_em_tc(cudaStream_t s, const float* X, int64_t n, int D, int K
 #ifdef FLASHGMM_DEBUG
     p.dbg = g_tc_debug;
     p.dbg_clk = g_tc_clk;
+    p.dbg_trace = g_tc_trace;
 #endif
     cudaError_t e = cudaFuncSetAttribute(em_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e != cudaSuccess) return e;

@@ -341,6 +341,7 @@ int gmm_create(gmm_ctx** out, int device, void* cuda_stream) {
     ctx->stream = static_cast<cudaStream_t>(cuda_stream);
     if (const char* e = std::getenv("GMM_TC_COND_LIMIT")) ctx->tc_cond_limit = (float)std::atof(e);
     if (const char* e = std::getenv("GMM_TC_FLUSH")) ctx->tc_flush = std::atoi(e);
+    if (const char* e = std::getenv("GMM_TC_ORDER")) tc_set_order(std::atoi(e));
     *out = ctx;
     return GMM_OK;
 }

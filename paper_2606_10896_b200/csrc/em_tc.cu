@@ -309,7 +309,7 @@ struct TcKernelParams {
     double* partial;               // [Q][TC_PCOLS][CL*128]  (+=)
     double* llpart;                // [2 Q]
     XSlot* xg;                     // [Q][4][CL][64] exchange slots (zeroed before every launch)
-    XSlot* xl;                     // [Q][4][CL][64] lower-bound exchange slots
+    XSlot* xl;                     // [Q][4][CL][4][64] lower-bound slots, one per warp and point
     int* status;
 #ifdef FLASHGMM_DEBUG
     float* dbg;      // [Kpad][64] log2 z of the first tile
@@ -400,11 +400,14 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
         const float ck = p.ck[rank * 128 + kloc];
         const float illb = p.illb[rank * 128 + kloc];
         const bool any_ill = p.flags[0] != 0;
+        float emax_w = illb;                                    // largest error bound among this warp's components
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) emax_w = fmaxf(emax_w, __shfl_xor_sync(0xffffffffu, emax_w, o));
         float* gather = reinterpret_cast<float*>(smem + SM_GATHER) + warp * 32;    // [8 warps][32]
         float2* ws = reinterpret_cast<float2*>(smem + SM_WS) + grp * 128;          // [4][32] per group
         float* fac = reinterpret_cast<float*>(smem + SM_FAC) + grp * 128;          // [4][32] per group
         XSlot* xg = p.xg + (size_t)cluster_id * 4 * p.CL * 64;             // [4][CL][64] ring of exchange slots
-        XSlot* xl = p.xl + (size_t)cluster_id * 4 * p.CL * 64;             // same, for the lower-bound exchange
+        XSlot* xl = p.xl + (size_t)cluster_id * 4 * p.CL * 256;            // [4][CL][4 warps][64]: lower bounds (ill-conditioned mode)
         float nk_acc = 0.f;
         double ll_acc = 0.0;
         // partial layout [group][column][component]: the 32 lanes of a warp touch 32 consecutive doubles; every address
@@ -442,75 +445,80 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
             TOC(tk_, 16);
             float red;
             // Ill-conditioned components (sum_d mu^2 / var too large for the 22-bit expanded form, e.g. a component
-            // collapsed onto a few points): their approximate logits carry an error of up to E_k.  A (component, point)
-            // pair can only matter if its upper bound l + E_k reaches the best LOWER bound max_k' (l - E_k') over ALL K
-            // components minus the 2^-40 margin, so the lower bounds are maximised over the group first (one extra
-            // exchange, only in launches that have such components).  Pairs that pass are recomputed exactly with
-            // direct differences in fp32, the whole warp working on one pair at a time; the rest are provably negligible.
+            // collapsed onto one point at the variance floor): their approximate logits carry an error of up to E_k.
+            // A (component, point) pair can only matter if its upper bound l + E_k reaches the best LOWER bound
+            // max_k' (l - E_k') over ALL K components minus the 2^-40 margin.  In launches that have such components
+            // every warp publishes a lower bound of its per-point maximum (a store, no wait, no barrier).  A warp first tests its
+            // flagged lanes against the warp's own bound (a weaker, local bound that already discards
+            // almost everything: a collapsed component is hopeless for every point but its own); the rare survivors
+            // are checked against the group-wide bound read from the published slots and, if they pass, recomputed
+            // exactly with direct differences in fp32, the whole warp working on one pair at a time.
+            // warp-level max per point (lane j ends up with point j)
+            warp_reduce_scatter32<true>(l, red, lane);
             if (any_ill) {
-                float* lbw = reinterpret_cast<float*>(smem + SM_LBW) + grp * 128;       // [4][32]
-                float* lbg = reinterpret_cast<float*>(smem + SM_LBG) + grp * 32;        // [32]
-                if (illb > 0.f) {
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) l[j] -= illb;
-                }
-                warp_reduce_scatter32<true>(l, red, lane);
-                if (illb > 0.f) {
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) l[j] += illb;      // (restores l up to ulp(E_k): irrelevant next to E_k)
-                }
-                lbw[wq * 32 + lane] = red;
-                named_bar_sync(7 + 2 * grp, 128);
-                if (gtid < 32) {
-                    const float m4 = fmaxf(fmaxf(lbw[gtid], lbw[32 + gtid]), fmaxf(lbw[64 + gtid], lbw[96 + gtid]));
-                    const uint32_t tag = (uint32_t)(i + 1);
-                    XSlot* ring = xl + (size_t)(i & 3) * p.CL * 64 + p0 + gtid;
-                    xslot_write(ring + rank * 64, m4, 0.f, tag);
-                    float2 e[8];
-                    if (!xslot_wait_all(ring, p.CL, tag, e, abort_flag, p.status)) alive = false;
-                    float mg = -CUDART_INF_F;
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) mg = fmaxf(mg, e[c].x);
-                    lbg[gtid] = mg;
-                }
-                named_bar_sync(8 + 2 * grp, 128);
-                if (__any_sync(0xffffffffu, illb > 0.f)) {
+                // max_k (l_k - E_k) >= max_k l_k - max_k E_k: the warp maximum minus the warp's largest error bound is a
+                // valid lower bound (and for a warp without flagged lanes it is the maximum itself)
+                const uint32_t tag = (uint32_t)(i + 1);
+                XSlot* ring = xl + (size_t)(i & 3) * p.CL * 256 + p0;
+                xslot_write(ring + (rank * 4 + wq) * 64 + lane, red - emax_w, 0.f, tag);     // publish: no barrier, no wait
+                if (emax_w > 0.f) {
+                    gather[lane] = red - emax_w;
+                    __syncwarp();
                     const int kglob = (int)rank * 128 + kloc;
                     uint32_t mlo = 0;
                     if (illb > 0.f) {
 #pragma unroll
                         for (int j = 0; j < 32; ++j)
-                            if (j < nvalid && l[j] + illb >= lbg[j] - ILL_MARGIN) mlo |= 1u << j;
+                            if (j < nvalid && l[j] + illb >= gather[j] - ILL_MARGIN) mlo |= 1u << j;
                     }
+                    bool fixed_any = false;
                     for (;;) {
                         const uint32_t ballot = __ballot_sync(0xffffffffu, mlo != 0u);
                         if (ballot == 0u) break;
                         const int src = __ffs(ballot) - 1;
                         int j = __ffs(mlo) - 1;
-                        j = __shfl_sync(0xffffffffu, j, src);
-                        const int kk = __shfl_sync(0xffffffffu, kglob, src);
-                        const float* xr = p.X + (row0 + p0 + j) * p.D;
-                        const float* mr = p.mu + (size_t)kk * p.D;
-                        const float* wr = p.w2 + (size_t)kk * p.D;
-                        float q = 0.f;
-                        for (int d = lane; d < p.D; d += 32) {
-                            const float diff = __ldg(xr + d) - __ldg(mr + d);
-                            q = fmaf(diff * diff, __ldg(wr + d), q);
-                        }
-#pragma unroll
-                        for (int o = 16; o > 0; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
-                        const float val = __ldg(p.c2 + kk) - q;
+                        float ub = -CUDART_INF_F;                  // upper bound l + E of the owner's candidate
                         if (lane == src) {
 #pragma unroll
                             for (int jj = 0; jj < 32; ++jj)
-                                if (jj == j) l[jj] = val;
-                            mlo &= ~(1u << j);
+                                if (jj == j) ub = l[jj] + illb;
                         }
+                        j = __shfl_sync(0xffffffffu, j, src);
+                        ub = __shfl_sync(0xffffffffu, ub, src);
+                        const int kk = __shfl_sync(0xffffffffu, kglob, src);
+                        // group-wide lower-bound maximum of point j: lane c reads the slot of (CTA c / 4, warp c % 4)
+                        float lbv = -CUDART_INF_F, dummy = 0.f;
+                        if (lane < 4 * p.CL) {
+                            if (!xslot_wait(ring + lane * 64 + j, tag, lbv, dummy, abort_flag, p.status)) alive = false;
+                        }
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) lbv = fmaxf(lbv, __shfl_xor_sync(0xffffffffu, lbv, o));
+                        if (ub >= lbv - ILL_MARGIN) {
+                            const float* xr = p.X + (row0 + p0 + j) * p.D;
+                            const float* mr = p.mu + (size_t)kk * p.D;
+                            const float* wr = p.w2 + (size_t)kk * p.D;
+                            float q = 0.f;
+                            for (int d = lane; d < p.D; d += 32) {
+                                const float diff = __ldg(xr + d) - __ldg(mr + d);
+                                q = fmaf(diff * diff, __ldg(wr + d), q);
+                            }
+#pragma unroll
+                            for (int o = 16; o > 0; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
+                            const float val = __ldg(p.c2 + kk) - q;
+                            if (lane == src) {
+#pragma unroll
+                                for (int jj = 0; jj < 32; ++jj)
+                                    if (jj == j) l[jj] = val;
+                            }
+                            fixed_any = true;
+                        }
+                        if (lane == src) mlo &= ~(1u << j);
                     }
+                    __syncwarp();
+                    if (fixed_any) warp_reduce_scatter32<true>(l, red, lane);      // maxima with the corrected logits
                 }
             }
-            // warp-level max per point (lane j ends up with point j), all-gathered through shared memory
-            warp_reduce_scatter32<true>(l, red, lane);
+            // all-gather the warp maxima through shared memory
             gather[lane] = red;
             __syncwarp();
             TOC(tk_, 17);
@@ -1030,7 +1038,7 @@ size_t tc_scratch_bytes(int D, int K) {
     b += (size_t)pl.Kpad * 4 * 2 + 512;                    // t_k, c_k, s_d
     b += (size_t)pl.Q * pl.Kpad * TC_PCOLS * 8;            // float64 partials
     b += (size_t)pl.Q * 16;
-    b += 2 * (size_t)pl.Q * 4 * pl.CL * 64 * 16;           // exchange slots
+    b += 5 * (size_t)pl.Q * 4 * pl.CL * 64 * 16;           // exchange slots
     return b + 8 * 256;
 }
 
@@ -1069,7 +1077,7 @@ cudaError_t launch_em_tc(cudaStream_t s, const float* X, int64_t n, int D, int K
     const size_t xbytes = (size_t)Q * 4 * pl.CL * 64 * sizeof(XSlot);
     e = cudaMemsetAsync(tb.xg, 0, xbytes, s);
     if (e != cudaSuccess) return e;
-    e = cudaMemsetAsync(tb.xl, 0, xbytes, s);
+    e = cudaMemsetAsync(tb.xl, 0, 4 * xbytes, s);
     if (e != cudaSuccess) return e;
     // The CTAs of a group wait for one another, so all of them must be resident at once: a cooperative launch either
     // guarantees that or fails.

@@ -58,7 +58,7 @@ ScratchLayout scratch_layout(int D, int K) {
         L.tc_illb = take((size_t)pl.Kpad * 4);
         L.tc_flags = take(16);
         L.tc_xg = take((size_t)pl.Q * 4 * pl.CL * 64 * 16);
-        L.tc_xl = take((size_t)pl.Q * 4 * pl.CL * 64 * 16);
+        L.tc_xl = take((size_t)pl.Q * 4 * pl.CL * 256 * 16);
         L.tc_partial_bytes = (size_t)pl.Q * pl.Kpad * TC_PCOLS * 8;
         L.tc_partial = take(L.tc_partial_bytes);
         L.tc_llpart = take((size_t)pl.Q * 16);

@@ -35,14 +35,19 @@ __device__ __forceinline__ float fast_ex2(float x) {
 
 // q[a][b] = sum_d w2[k0 + 4 tx + b][d] * (X[row0 + 4 ty + a][d] - mu[k0 + 4 tx + b][d])^2
 // Rows >= n and components >= K are staged as zeros (w2 = 0 -> contributes nothing).
+// ACC = float: one fp32 accumulation chain over D (D <= 128: a few 1e-6 of error).  ACC = double: each 32-dimension
+// chunk is summed in fp32 and the chunk sums are added in float64, which keeps long chains (D = 768: |q| ~ 1000 in the
+// log2 domain) from drowning the responsibilities in rounding noise.
+template <typename ACC>
 __device__ __forceinline__ void tile_quadratic(TileSmem& sm, const float* __restrict__ X, int64_t row0, int64_t n,
                                                int D, const float* __restrict__ mu, const float* __restrict__ w2,
-                                               int k0, int K, float (&q)[4][4]) {
+                                               int k0, int K, ACC (&q)[4][4]) {
+    constexpr bool HP = sizeof(ACC) == 8;
     const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
 #pragma unroll
     for (int a = 0; a < 4; ++a)
 #pragma unroll
-        for (int b = 0; b < 4; ++b) q[a][b] = 0.f;
+        for (int b = 0; b < 4; ++b) q[a][b] = (ACC)0;
     for (int d0 = 0; d0 < D; d0 += DCH) {
         __syncthreads();
 #pragma unroll
@@ -63,6 +68,11 @@ __device__ __forceinline__ void tile_quadratic(TileSmem& sm, const float* __rest
             sm.ws[c][r] = wv;
         }
         __syncthreads();
+        float part[4][4];
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+#pragma unroll
+            for (int b = 0; b < 4; ++b) part[a][b] = HP ? 0.f : (float)q[a][b];
 #pragma unroll 8
         for (int c = 0; c < DCH; ++c) {
             const float4 xv = *reinterpret_cast<const float4*>(&sm.xs[c][4 * ty]);
@@ -76,29 +86,33 @@ __device__ __forceinline__ void tile_quadratic(TileSmem& sm, const float* __rest
 #pragma unroll
                 for (int b = 0; b < 4; ++b) {
                     const float diff = xa[a] - mb[b];
-                    q[a][b] = fmaf(diff * diff, wb[b], q[a][b]);
+                    part[a][b] = fmaf(diff * diff, wb[b], part[a][b]);
                 }
         }
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+#pragma unroll
+            for (int b = 0; b < 4; ++b) q[a][b] = HP ? (ACC)(q[a][b] + (ACC)part[a][b]) : (ACC)part[a][b];
     }
 }
 
-template <int M>
+template <int M, typename ACC>
 struct TopList {
-    float v[M];
+    ACC v[M];
     int i[M];
     __device__ __forceinline__ void init() {
 #pragma unroll
-        for (int j = 0; j < M; ++j) { v[j] = -CUDART_INF_F; i[j] = -1; }
+        for (int j = 0; j < M; ++j) { v[j] = (ACC)(-CUDART_INF_F); i[j] = -1; }
     }
     // insert keeping descending order; equal values keep the earlier (smaller) index first
-    __device__ __forceinline__ void insert(float val, int id) {
+    __device__ __forceinline__ void insert(ACC val, int id) {
         if (i[M - 1] >= 0 && !(val > v[M - 1])) return;
         v[M - 1] = val; i[M - 1] = id;
 #pragma unroll
         for (int j = M - 1; j > 0; --j) {
             const bool up = (i[j - 1] < 0) || (v[j] > v[j - 1]);
             if (up) {
-                const float tv = v[j]; v[j] = v[j - 1]; v[j - 1] = tv;
+                const ACC tv = v[j]; v[j] = v[j - 1]; v[j - 1] = tv;
                 const int ti = i[j]; i[j] = i[j - 1]; i[j - 1] = ti;
             }
         }
@@ -106,38 +120,42 @@ struct TopList {
 };
 
 // M == 0: log-sum-exp only.  M > 0: also the top-M components per point.
-template <int M>
+// ACC is the type the logits are carried in: float for D <= 128, double beyond (see tile_quadratic).  The exponentials
+// always take a float argument formed AFTER the subtraction of the reference, so large common offsets cancel exactly.
+template <int M, typename ACC>
 __global__ void __launch_bounds__(NTHREADS)
 lse_kernel(const float* __restrict__ X, int64_t n, int D, int K, const float* __restrict__ mu,
-           const float* __restrict__ w2, const float* __restrict__ c2, float* __restrict__ logZ2,
+           const float* __restrict__ w2, const double* __restrict__ c2, double* __restrict__ logZ2,
            double* __restrict__ llpart, int m_out, int32_t* __restrict__ idx_out, float* __restrict__ resp_out) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     TileSmem& sm = *reinterpret_cast<TileSmem*>(smem_raw);
     __shared__ double ll_s[TP];
     const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
     const int64_t row0 = (int64_t)blockIdx.x * TP;
+    const ACC NEG_INF = (ACC)(-CUDART_INF_F);
 
-    float m_run[4], s_run[4];
+    ACC m_run[4];
+    float s_run[4];
 #pragma unroll
-    for (int a = 0; a < 4; ++a) { m_run[a] = -CUDART_INF_F; s_run[a] = 0.f; }
-    TopList<(M > 0 ? M : 1)> top[4];
+    for (int a = 0; a < 4; ++a) { m_run[a] = NEG_INF; s_run[a] = 0.f; }
+    TopList<(M > 0 ? M : 1), ACC> top[4];
     if (M > 0) {
 #pragma unroll
         for (int a = 0; a < 4; ++a) top[a].init();
     }
 
     for (int k0 = 0; k0 < K; k0 += TC) {
-        float q[4][4];
-        tile_quadratic(sm, X, row0, n, D, mu, w2, k0, K, q);
-        float cv[4];
+        ACC q[4][4];
+        tile_quadratic<ACC>(sm, X, row0, n, D, mu, w2, k0, K, q);
+        ACC cv[4];
 #pragma unroll
         for (int b = 0; b < 4; ++b) {
             const int k = k0 + 4 * tx + b;
-            cv[b] = (k < K) ? __ldg(c2 + k) : -CUDART_INF_F;
+            cv[b] = (k < K) ? (ACC)__ldg(c2 + k) : NEG_INF;
         }
 #pragma unroll
         for (int a = 0; a < 4; ++a) {
-            float l[4];
+            ACC l[4];
 #pragma unroll
             for (int b = 0; b < 4; ++b) l[b] = cv[b] - q[a][b];
             if (M > 0) {
@@ -145,37 +163,42 @@ lse_kernel(const float* __restrict__ X, int64_t n, int D, int K, const float* __
                 for (int b = 0; b < 4; ++b)
                     if (k0 + 4 * tx + b < K) top[a].insert(l[b], k0 + 4 * tx + b);
             }
-            float mloc = fmaxf(fmaxf(l[0], l[1]), fmaxf(l[2], l[3]));
+            ACC mloc = l[0] > l[1] ? l[0] : l[1];
+            mloc = l[2] > mloc ? l[2] : mloc;
+            mloc = l[3] > mloc ? l[3] : mloc;
 #pragma unroll
-            for (int o = 8; o > 0; o >>= 1) mloc = fmaxf(mloc, __shfl_xor_sync(0xffffffffu, mloc, o));
-            const float m_new = fmaxf(m_run[a], mloc);
-            const float m_safe = (m_new == -CUDART_INF_F) ? 0.f : m_new;
-            float sloc = fast_ex2(l[0] - m_safe) + fast_ex2(l[1] - m_safe) + fast_ex2(l[2] - m_safe) +
-                         fast_ex2(l[3] - m_safe);
+            for (int o = 8; o > 0; o >>= 1) {
+                const ACC other = __shfl_xor_sync(0xffffffffu, mloc, o);
+                mloc = other > mloc ? other : mloc;
+            }
+            const ACC m_new = m_run[a] > mloc ? m_run[a] : mloc;
+            const ACC m_safe = (m_new == NEG_INF) ? (ACC)0 : m_new;
+            float sloc = fast_ex2((float)(l[0] - m_safe)) + fast_ex2((float)(l[1] - m_safe)) +
+                         fast_ex2((float)(l[2] - m_safe)) + fast_ex2((float)(l[3] - m_safe));
 #pragma unroll
             for (int o = 8; o > 0; o >>= 1) sloc += __shfl_xor_sync(0xffffffffu, sloc, o);
-            s_run[a] = s_run[a] * fast_ex2(m_run[a] - m_safe) + sloc;
+            s_run[a] = s_run[a] * fast_ex2((float)(m_run[a] - m_safe)) + sloc;
             m_run[a] = m_new;
         }
     }
 
-    float lz[4];
+    double lz[4];
 #pragma unroll
-    for (int a = 0; a < 4; ++a) lz[a] = m_run[a] + log2f(s_run[a]);
+    for (int a = 0; a < 4; ++a) lz[a] = (double)m_run[a] + (double)log2f(s_run[a]);
     if (tx == 0) {
 #pragma unroll
         for (int a = 0; a < 4; ++a) {
             const int64_t row = row0 + 4 * ty + a;
             const bool ok = row < n;
             if (ok && logZ2) logZ2[row] = lz[a];
-            ll_s[4 * ty + a] = ok ? (double)lz[a] * 0.69314718055994530942 : 0.0;
+            ll_s[4 * ty + a] = ok ? lz[a] * 0.69314718055994530942 : 0.0;
         }
     }
     if (M > 0) {
         // merge the 16 per-thread lists of each point through shared memory (reuses the staging area)
         __syncthreads();
-        float* cand_v = reinterpret_cast<float*>(smem_raw);
-        int* cand_i = reinterpret_cast<int*>(smem_raw) + TP * 16 * M;
+        ACC* cand_v = reinterpret_cast<ACC*>(smem_raw);
+        int* cand_i = reinterpret_cast<int*>(cand_v + TP * 16 * M);
 #pragma unroll
         for (int a = 0; a < 4; ++a)
 #pragma unroll
@@ -184,16 +207,16 @@ lse_kernel(const float* __restrict__ X, int64_t n, int D, int K, const float* __
                 cand_v[slot] = top[a].v[j];
                 cand_i[slot] = top[a].i[j];
             }
-        __shared__ float lz_s[TP];
+        __shared__ double lz_s[TP];
         if (tx == 0) {
 #pragma unroll
             for (int a = 0; a < 4; ++a) lz_s[4 * ty + a] = lz[a];
         }
         __syncthreads();
         if (tid < TP && row0 + tid < n) {
-            float* cv = cand_v + tid * 16 * M;
+            ACC* cv = cand_v + tid * 16 * M;
             int* ci = cand_i + tid * 16 * M;
-            const float lzp = lz_s[tid];
+            const double lzp = lz_s[tid];
             for (int j = 0; j < m_out; ++j) {
                 int best = -1;
                 for (int s = 0; s < 16 * M; ++s) {
@@ -204,7 +227,7 @@ lse_kernel(const float* __restrict__ X, int64_t n, int D, int K, const float* __
                 float r = 0.f;
                 if (best >= 0) {
                     id = ci[best];
-                    r = fast_ex2(cv[best] - lzp);
+                    r = fast_ex2((float)((double)cv[best] - lzp));
                     ci[best] = -1;
                 }
                 idx_out[(row0 + tid) * m_out + j] = id;
@@ -226,9 +249,10 @@ constexpr int LDR = TC + 4;                 // r tile row stride
 constexpr int LDX = FP32_MSTEP_DC + 4;      // X tile row stride
 constexpr size_t MSTEP_SMEM = sizeof(TileSmem) + (size_t)TP * LDR * 4 + (size_t)TP * LDX * 4;
 
+template <typename ACC>
 __global__ void __launch_bounds__(NTHREADS)
 mstep_kernel(const float* __restrict__ X, int64_t n, int D, int K, const float* __restrict__ mu,
-             const float* __restrict__ w2, const float* __restrict__ c2, const float* __restrict__ logZ2,
+             const float* __restrict__ w2, const double* __restrict__ c2, const double* __restrict__ logZ2,
              float* __restrict__ partials) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     TileSmem& sm = *reinterpret_cast<TileSmem*>(smem_raw);
@@ -247,26 +271,26 @@ mstep_kernel(const float* __restrict__ X, int64_t n, int D, int K, const float* 
 #pragma unroll
         for (int j = 0; j < 4; ++j) { acc1[c][j] = 0.f; acc2[c][j] = 0.f; }
     float nacc = 0.f;
-    float cv[4];
+    ACC cv[4];
 #pragma unroll
     for (int b = 0; b < 4; ++b) {
         const int k = k0 + 4 * tx + b;
-        cv[b] = (k < K) ? __ldg(c2 + k) : -CUDART_INF_F;
+        cv[b] = (k < K) ? (ACC)__ldg(c2 + k) : (ACC)(-CUDART_INF_F);
     }
 
     for (int64_t t = split; t < ntiles; t += nsplits) {
         const int64_t row0 = t * TP;
-        float q[4][4];
-        tile_quadratic(sm, X, row0, n, D, mu, w2, k0, K, q);
+        ACC q[4][4];
+        tile_quadratic<ACC>(sm, X, row0, n, D, mu, w2, k0, K, q);
 #pragma unroll
         for (int a = 0; a < 4; ++a) {
             const int64_t row = row0 + 4 * ty + a;
-            const float lz = (row < n) ? __ldg(logZ2 + row) : CUDART_INF_F;    // +inf -> r = 0 for padded rows
+            const ACC lz = (row < n) ? (ACC)__ldg(logZ2 + row) : (ACC)CUDART_INF_F;    // +inf -> r = 0 for padded rows
             float4 rv;
-            rv.x = fast_ex2(cv[0] - q[a][0] - lz);
-            rv.y = fast_ex2(cv[1] - q[a][1] - lz);
-            rv.z = fast_ex2(cv[2] - q[a][2] - lz);
-            rv.w = fast_ex2(cv[3] - q[a][3] - lz);
+            rv.x = fast_ex2((float)(cv[0] - q[a][0] - lz));
+            rv.y = fast_ex2((float)(cv[1] - q[a][1] - lz));
+            rv.z = fast_ex2((float)(cv[2] - q[a][2] - lz));
+            rv.w = fast_ex2((float)(cv[3] - q[a][3] - lz));
             *reinterpret_cast<float4*>(&r_s[(4 * ty + a) * LDR + 4 * tx]) = rv;
         }
         // stage this CTA's D-slice of the X tile, row-major
@@ -326,7 +350,7 @@ mstep_kernel(const float* __restrict__ X, int64_t n, int D, int K, const float* 
 // One block per component: w2 = (log2 e / 2) / var, c2 = log2 e (log pi - 1/2 sum_d log(2 pi var)), in float64.
 __global__ void prepare_fp32_kernel(int D, int K, const float* __restrict__ pi, const float* __restrict__ mu,
                                     const float* __restrict__ var, float* __restrict__ w2, float* __restrict__ c2,
-                                    int* __restrict__ status) {
+                                    double* __restrict__ c2d, int* __restrict__ status) {
     const int k = blockIdx.x;
     __shared__ double red[128];
     double s = 0.0;
@@ -350,7 +374,9 @@ __global__ void prepare_fp32_kernel(int D, int K, const float* __restrict__ pi, 
         const float p = pi[k];
         if (!(p >= 0.f) || !isfinite(p)) bad |= ST_BAD_PI;
         const double lp = (p > 0.f) ? log((double)p) : -CUDART_INF;
-        c2[k] = (float)(1.4426950408889634074 * (lp - 0.5 * red[0]));
+        const double cd = 1.4426950408889634074 * (lp - 0.5 * red[0]);
+        c2[k] = (float)cd;
+        c2d[k] = cd;
     }
     if (bad) atomicOr(status, bad);
 }
@@ -373,47 +399,64 @@ size_t fp32_partial_floats(int D, int K) {
 }
 
 cudaError_t launch_prepare_fp32(cudaStream_t s, int D, int K, const float* pi, const float* mu, const float* var,
-                                float* w2, float* c2, int* status) {
-    prepare_fp32_kernel<<<K, 128, 0, s>>>(D, K, pi, mu, var, w2, c2, status);
+                                float* w2, float* c2, double* c2d, int* status) {
+    prepare_fp32_kernel<<<K, 128, 0, s>>>(D, K, pi, mu, var, w2, c2, c2d, status);
     return cudaGetLastError();
 }
+
+// Logits are carried in float64 when the accumulation over D is long.
+static inline bool fp32_high_precision(int D) { return D > 128; }
 
 cudaError_t launch_lse_fp32(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu,
-                            const float* w2, const float* c2, float* logZ2, double* llpart) {
+                            const float* w2, const double* c2d, double* logZ2, double* llpart) {
     const unsigned blocks = (unsigned)((n + TP - 1) / TP);
-    lse_kernel<0><<<blocks, NTHREADS, sizeof(TileSmem), s>>>(X, n, D, K, mu, w2, c2, logZ2, llpart, 0, nullptr,
-                                                            nullptr);
+    if (fp32_high_precision(D))
+        lse_kernel<0, double><<<blocks, NTHREADS, sizeof(TileSmem), s>>>(X, n, D, K, mu, w2, c2d, logZ2, llpart, 0, nullptr, nullptr);
+    else
+        lse_kernel<0, float><<<blocks, NTHREADS, sizeof(TileSmem), s>>>(X, n, D, K, mu, w2, c2d, logZ2, llpart, 0, nullptr, nullptr);
     return cudaGetLastError();
 }
 
-template <int M>
+template <int M, typename ACC>
 static cudaError_t launch_topm_t(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu,
-                                 const float* w2, const float* c2, int m, int32_t* idx, float* resp) {
+                                 const float* w2, const double* c2d, int m, int32_t* idx, float* resp) {
     size_t smem = sizeof(TileSmem);
-    const size_t need = (size_t)TP * 16 * M * 8;
+    const size_t need = (size_t)TP * 16 * M * (sizeof(ACC) + 4);
     if (need > smem) smem = need;
-    cudaError_t e = cudaFuncSetAttribute(lse_kernel<M>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(lse_kernel<M, ACC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     const unsigned blocks = (unsigned)((n + TP - 1) / TP);
-    lse_kernel<M><<<blocks, NTHREADS, smem, s>>>(X, n, D, K, mu, w2, c2, nullptr, nullptr, m, idx, resp);
+    lse_kernel<M, ACC><<<blocks, NTHREADS, smem, s>>>(X, n, D, K, mu, w2, c2d, nullptr, nullptr, m, idx, resp);
     return cudaGetLastError();
 }
 
 cudaError_t launch_topm_fp32(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu,
-                             const float* w2, const float* c2, int m, int32_t* idx, float* resp) {
-    if (m <= 1) return launch_topm_t<1>(s, X, n, D, K, mu, w2, c2, m, idx, resp);
-    if (m <= 2) return launch_topm_t<2>(s, X, n, D, K, mu, w2, c2, m, idx, resp);
-    if (m <= 4) return launch_topm_t<4>(s, X, n, D, K, mu, w2, c2, m, idx, resp);
-    return launch_topm_t<8>(s, X, n, D, K, mu, w2, c2, m, idx, resp);
+                             const float* w2, const double* c2d, int m, int32_t* idx, float* resp) {
+    if (fp32_high_precision(D)) {
+        if (m <= 1) return launch_topm_t<1, double>(s, X, n, D, K, mu, w2, c2d, m, idx, resp);
+        if (m <= 2) return launch_topm_t<2, double>(s, X, n, D, K, mu, w2, c2d, m, idx, resp);
+        if (m <= 4) return launch_topm_t<4, double>(s, X, n, D, K, mu, w2, c2d, m, idx, resp);
+        return launch_topm_t<8, double>(s, X, n, D, K, mu, w2, c2d, m, idx, resp);
+    }
+    if (m <= 1) return launch_topm_t<1, float>(s, X, n, D, K, mu, w2, c2d, m, idx, resp);
+    if (m <= 2) return launch_topm_t<2, float>(s, X, n, D, K, mu, w2, c2d, m, idx, resp);
+    if (m <= 4) return launch_topm_t<4, float>(s, X, n, D, K, mu, w2, c2d, m, idx, resp);
+    return launch_topm_t<8, float>(s, X, n, D, K, mu, w2, c2d, m, idx, resp);
 }
 
 cudaError_t launch_mstep_fp32(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu,
-                              const float* w2, const float* c2, const float* logZ2, float* partials,
+                              const float* w2, const double* c2d, const double* logZ2, float* partials,
                               const Fp32Plan& plan) {
-    cudaError_t e = cudaFuncSetAttribute(mstep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)MSTEP_SMEM);
-    if (e != cudaSuccess) return e;
     dim3 grid(plan.comp_blocks, plan.splits, plan.d_chunks);
-    mstep_kernel<<<grid, NTHREADS, MSTEP_SMEM, s>>>(X, n, D, K, mu, w2, c2, logZ2, partials);
+    if (fp32_high_precision(D)) {
+        cudaError_t e = cudaFuncSetAttribute(mstep_kernel<double>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)MSTEP_SMEM);
+        if (e != cudaSuccess) return e;
+        mstep_kernel<double><<<grid, NTHREADS, MSTEP_SMEM, s>>>(X, n, D, K, mu, w2, c2d, logZ2, partials);
+    } else {
+        cudaError_t e = cudaFuncSetAttribute(mstep_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)MSTEP_SMEM);
+        if (e != cudaSuccess) return e;
+        mstep_kernel<float><<<grid, NTHREADS, MSTEP_SMEM, s>>>(X, n, D, K, mu, w2, c2d, logZ2, partials);
+    }
     return cudaGetLastError();
 }
 

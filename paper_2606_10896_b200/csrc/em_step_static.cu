@@ -31,7 +31,7 @@ struct StaticResult {
 };
 
 struct StaticLayout {
-    size_t w2, c2, logZ2, llpart, result, partials, total;
+    size_t w2, c2, c2d, logZ2, llpart, result, partials, total;
     int splits;
 };
 
@@ -46,7 +46,8 @@ StaticLayout static_layout(int D, int K) {
     auto take = [&](size_t bytes) { size_t o = off; off += al(bytes); return o; };
     L.w2 = take(KD * 4);
     L.c2 = take((size_t)K * 4);
-    L.logZ2 = take((size_t)STATIC_TILE * 4);
+    L.c2d = take((size_t)K * 8);
+    L.logZ2 = take((size_t)STATIC_TILE * 8);
     L.llpart = take((size_t)(STATIC_TILE / FP32_TILE_P) * 8);
     L.result = take(sizeof(StaticResult));
     L.partials = take((size_t)L.splits * ((size_t)K + 2 * KD) * 4);
@@ -101,7 +102,8 @@ extern "C" int gmm_em_step_static(int device, void* cuda_stream, const float* X,
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     float* w2 = reinterpret_cast<float*>(base + L.w2);
     float* c2 = reinterpret_cast<float*>(base + L.c2);
-    float* logZ2 = reinterpret_cast<float*>(base + L.logZ2);
+    double* c2d = reinterpret_cast<double*>(base + L.c2d);
+    double* logZ2 = reinterpret_cast<double*>(base + L.logZ2);
     double* llpart = reinterpret_cast<double*>(base + L.llpart);
     StaticResult* res = reinterpret_cast<StaticResult*>(base + L.result);
     float* partials = reinterpret_cast<float*>(base + L.partials);
@@ -115,12 +117,12 @@ extern "C" int gmm_em_step_static(int device, void* cuda_stream, const float* X,
     SCU(cudaMemsetAsync(Nk, 0, (size_t)K * 8, s));
     SCU(cudaMemsetAsync(S1, 0, KD * 8, s));
     SCU(cudaMemsetAsync(S2, 0, KD * 8, s));
-    SCU(launch_prepare_fp32(s, D, K, pi, mu, var, w2, c2, &res->status));
+    SCU(launch_prepare_fp32(s, D, K, pi, mu, var, w2, c2, c2d, &res->status));
     for (int64_t off = 0; off < N; off += STATIC_TILE) {
         const int64_t cnt = (N - off < STATIC_TILE) ? (N - off) : STATIC_TILE;
         const float* Xs = X + off * D;
-        SCU(launch_lse_fp32(s, Xs, cnt, D, K, mu, w2, c2, logZ2, llpart));
-        SCU(launch_mstep_fp32(s, Xs, cnt, D, K, mu, w2, c2, logZ2, partials, plan));
+        SCU(launch_lse_fp32(s, Xs, cnt, D, K, mu, w2, c2d, logZ2, llpart));
+        SCU(launch_mstep_fp32(s, Xs, cnt, D, K, mu, w2, c2d, logZ2, partials, plan));
         SCU(launch_reduce_ll(s, llpart, (cnt + FP32_TILE_P - 1) / FP32_TILE_P, &res->ll, true));
         SCU(launch_reduce_partials(s, D, K, plan.splits, partials, Nk, S1, S2, true));
     }

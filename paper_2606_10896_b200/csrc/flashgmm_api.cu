@@ -27,7 +27,7 @@ constexpr int EVENT_POOL = 128;
 inline size_t align256(size_t b) { return (b + 255) & ~(size_t)255; }
 
 struct ScratchLayout {
-    size_t w2, c2, partials, logZ2, llpart, result, stats, total;
+    size_t w2, c2, c2d, partials, logZ2, llpart, result, stats, total;
     size_t tc_phi, tc_plo, tc_tk, tc_ck, tc_sd, tc_kap, tc_illb, tc_flags, tc_xg, tc_xl, tc_partial, tc_llpart, tc_partial_bytes;
     bool tc;
 };
@@ -39,8 +39,9 @@ ScratchLayout scratch_layout(int D, int K) {
     auto take = [&](size_t bytes) { size_t o = off; off += align256(bytes); return o; };
     L.w2 = take(KD * 4);
     L.c2 = take((size_t)K * 4);
+    L.c2d = take((size_t)K * 8);
     L.partials = take(fp32_partial_floats(D, K) * 4);
-    L.logZ2 = take((size_t)SUPER_TILE * 4);
+    L.logZ2 = take((size_t)SUPER_TILE * 8);
     L.llpart = take((size_t)(SUPER_TILE / FP32_TILE_P) * 8);
     L.result = take(sizeof(DevResult));
     L.stats = take(((size_t)K + 2 * KD) * 8);
@@ -101,8 +102,9 @@ struct gmm_ctx {
 
     float* w2() const { return reinterpret_cast<float*>(scratch + lay.w2); }
     float* c2() const { return reinterpret_cast<float*>(scratch + lay.c2); }
+    double* c2d() const { return reinterpret_cast<double*>(scratch + lay.c2d); }
     float* partials() const { return reinterpret_cast<float*>(scratch + lay.partials); }
-    float* logZ2() const { return reinterpret_cast<float*>(scratch + lay.logZ2); }
+    double* logZ2() const { return reinterpret_cast<double*>(scratch + lay.logZ2); }
     double* llpart() const { return reinterpret_cast<double*>(scratch + lay.llpart); }
     DevResult* result() const { return reinterpret_cast<DevResult*>(scratch + lay.result); }
     double* stats() const { return reinterpret_cast<double*>(scratch + lay.stats); }
@@ -238,7 +240,7 @@ int prof_end(gmm_ctx* ctx) {
 int prepare_and_choose(gmm_ctx* ctx, int64_t N, int D, int K, const float* pi, const float* mu, const float* var,
                        int* path) {
     CU(cudaMemsetAsync(&ctx->result()->status, 0, sizeof(int), ctx->stream));
-    KL(launch_prepare_fp32(ctx->stream, D, K, pi, mu, var, ctx->w2(), ctx->c2(), &ctx->result()->status));
+    KL(launch_prepare_fp32(ctx->stream, D, K, pi, mu, var, ctx->w2(), ctx->c2(), ctx->c2d(), &ctx->result()->status));
     const bool tc_ok = ctx->lay.tc && ctx->tc_Q >= 1;
     const bool tc_auto = tc_ok && gmm_auto_path(D, K) == GMM_PATH_TENSOR;
     if (ctx->path == GMM_PATH_TENSOR && !tc_ok)
@@ -279,8 +281,8 @@ int accumulate_points(gmm_ctx* ctx, int path, const float* X, int64_t n, int D, 
         const int64_t cnt = (n - off < SUPER_TILE) ? (n - off) : SUPER_TILE;
         const float* Xs = X + off * D;
         CHECK(prof_begin(ctx));
-        KL(launch_lse_fp32(ctx->stream, Xs, cnt, D, K, mu, ctx->w2(), ctx->c2(), ctx->logZ2(), ctx->llpart()));
-        KL(launch_mstep_fp32(ctx->stream, Xs, cnt, D, K, mu, ctx->w2(), ctx->c2(), ctx->logZ2(), ctx->partials(), plan));
+        KL(launch_lse_fp32(ctx->stream, Xs, cnt, D, K, mu, ctx->w2(), ctx->c2d(), ctx->logZ2(), ctx->llpart()));
+        KL(launch_mstep_fp32(ctx->stream, Xs, cnt, D, K, mu, ctx->w2(), ctx->c2d(), ctx->logZ2(), ctx->partials(), plan));
         CHECK(prof_end(ctx));
         KL(launch_reduce_ll(ctx->stream, ctx->llpart(), (cnt + FP32_TILE_P - 1) / FP32_TILE_P, &ctx->result()->ll[slot], true));
         KL(launch_reduce_partials(ctx->stream, D, K, plan.splits, ctx->partials(), Nk, S1, S2, true));
@@ -544,10 +546,10 @@ int gmm_assign_topm(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const
     DeviceGuard g(ctx->device);
     CHECK(ensure_scratch(ctx, D, K));
     CU(cudaMemsetAsync(&ctx->result()->status, 0, sizeof(int), ctx->stream));
-    KL(launch_prepare_fp32(ctx->stream, D, K, pi, mu, var, ctx->w2(), ctx->c2(), &ctx->result()->status));
+    KL(launch_prepare_fp32(ctx->stream, D, K, pi, mu, var, ctx->w2(), ctx->c2(), ctx->c2d(), &ctx->result()->status));
     for (int64_t off = 0; off < N; off += SUPER_TILE) {
         const int64_t cnt = (N - off < SUPER_TILE) ? (N - off) : SUPER_TILE;
-        KL(launch_topm_fp32(ctx->stream, X + off * D, cnt, D, K, mu, ctx->w2(), ctx->c2(), m, idx + off * m, resp + off * m));
+        KL(launch_topm_fp32(ctx->stream, X + off * D, cnt, D, K, mu, ctx->w2(), ctx->c2d(), m, idx + off * m, resp + off * m));
     }
     ctx->last_path = GMM_PATH_FP32;
     return GMM_OK;

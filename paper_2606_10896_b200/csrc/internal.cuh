@@ -27,15 +27,16 @@ size_t fp32_partial_floats(int D, int K);   // floats in the per-CTA partial buf
 
 // ---- FP32 (CUDA-core) path -----------------------------------------------------------------------------------
 cudaError_t launch_prepare_fp32(cudaStream_t s, int D, int K, const float* pi, const float* mu, const float* var,
-                                float* w2, float* c2, int* status);
+                                float* w2, float* c2, double* c2d, int* status);
 // log2-domain log Z of n points -> logZ2[n]; per-block float64 partial log-likelihoods -> llpart[ceil(n/64)]
+// c2d: the per-component constants in float64; logZ2: float64 (the kernels carry logits in float64 when D > 128)
 cudaError_t launch_lse_fp32(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu,
-                            const float* w2, const float* c2, float* logZ2, double* llpart);
+                            const float* w2, const double* c2d, double* logZ2, double* llpart);
 cudaError_t launch_mstep_fp32(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu,
-                              const float* w2, const float* c2, const float* logZ2, float* partials,
+                              const float* w2, const double* c2d, const double* logZ2, float* partials,
                               const Fp32Plan& plan);
 cudaError_t launch_topm_fp32(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu,
-                             const float* w2, const float* c2, int m, int32_t* idx, float* resp);
+                             const float* w2, const double* c2d, int m, int32_t* idx, float* resp);
 
 // ---- shared by all paths -------------------------------------------------------------------------------------
 // stats (+)= sum over `splits` partial blocks, fixed order, float64.  Partial layout: [splits][K + 2*K*D] floats,

@@ -339,3 +339,92 @@ def test_config3_full_size_conservation_and_subsample(fg, ctx):
         got = _gpu_step(ctx, Xsub_d, pi0, mu0, var0)
         assert abs(got[3] - ref[3]) <= 1e-5 * abs(ref[3])
         assert_stats_close(len(rows), s, got[:3], ref[:3], f"path {path} config 3 subsample")
+
+
+def _column_sums(X):
+    """Column sums of X and X^2 in float64, in chunks (X may be tens of GB)."""
+    s1 = torch.zeros(X.shape[1], dtype=torch.float64, device=X.device)
+    s2 = torch.zeros_like(s1)
+    step = 1 << 22
+    for lo in range(0, X.shape[0], step):
+        x = X[lo:lo + step].double()
+        s1 += x.sum(0)
+        s2 += (x * x).sum(0)
+    return s1.cpu().numpy(), s2.cpu().numpy()
+
+
+def test_config4_full_size_conservation_additivity_and_subsample(fg, ctx):
+    """N = 100M, K = 1024, D = 128 (51.2 GB of X) in the launch configuration the benchmark times (AUTO path = the
+    tensor-core kernel): the conservation laws hold at full N, the statistics of the whole equal the sum over two
+    halves (long accumulation chains), device memory in use does not grow with N, and one oracle step on a seeded
+    50K-row subsample matches the GPU on the same rows."""
+    spec = synth.CONFIGS[4]
+    free_b, _ = torch.cuda.mem_get_info()
+    if free_b < 60e9:
+        pytest.skip("needs 60 GB of free device memory")
+    X = synth.sample_device(spec, DEV)
+    pi0, mu0, var0 = synth.init_params(X, spec)
+    N = spec.N
+    col1, col2 = _column_sums(X)
+    ctx.gmm_set_path(fg.GMM_PATH_AUTO)
+    torch.cuda.synchronize()
+    Nk, S1, S2, L = _gpu_step(ctx, X, pi0, mu0, var0)
+    assert ctx.gmm_last_path() == fg.GMM_PATH_TENSOR
+    free_after = torch.cuda.mem_get_info()[0]
+    s = float(np.sqrt(synth.global_variance(X[:1_000_000]).mean()))
+    assert abs(Nk.sum() - N) <= 1e-6 * N
+    np.testing.assert_allclose(S1.sum(0), col1, rtol=1e-5, atol=1e-5 * N * s)
+    np.testing.assert_allclose(S2.sum(0), col2, rtol=1e-5)
+    assert np.isfinite(L)
+    # additivity over two halves
+    h = N // 2
+    a = _gpu_step(ctx, X[:h], pi0, mu0, var0)
+    b = _gpu_step(ctx, X[h:], pi0, mu0, var0)
+    assert torch.cuda.mem_get_info()[0] == free_after, "device memory in use changed with N"
+    np.testing.assert_allclose(a[0] + b[0], Nk, rtol=1e-6, atol=1e-6 * N / spec.K)
+    np.testing.assert_allclose(a[2] + b[2], S2, rtol=2e-5, atol=1e-5 * N / spec.K)
+    assert abs((a[3] + b[3]) - L) <= 1e-9 * abs(L)
+    # oracle on a seeded subsample, GPU re-run on the same rows
+    rows = synth.subsample_rows(N, 50_000, spec.seed)
+    Xsub_d = X[torch.as_tensor(rows, device=DEV)].contiguous()
+    del X
+    Xsub = Xsub_d.cpu().numpy()
+    ref = orc.em_step(Xsub, pi0, mu0, var0)
+    got = _gpu_step(ctx, Xsub_d, pi0, mu0, var0)
+    assert abs(got[3] - ref[3]) <= 1e-5 * abs(ref[3])
+    assert_stats_close(len(rows), data_scale(Xsub), got[:3], ref[:3], "config 4 subsample")
+
+
+def test_config5_shape_step_and_topm_on_subsample(fg, ctx):
+    """The IVF coarse-quantizer shape (D = 768, K = 4096, unit-norm vectors): one EM step and top-4 assignment on
+    1M device-generated points (AUTO path = the FP32 kernels: the shape is outside the tensor path), conservation at
+    that N, and the oracle on a seeded 20K-row subsample for both the step and the top-4 output."""
+    spec = synth.CONFIGS[5].with_n(1_000_000)
+    X = synth.sample_device(spec, DEV)
+    pi0, mu0, var0 = synth.init_params(X, spec)
+    N = spec.N
+    col1, col2 = _column_sums(X)
+    ctx.gmm_set_path(fg.GMM_PATH_AUTO)
+    Nk, S1, S2, L = _gpu_step(ctx, X, pi0, mu0, var0)
+    assert ctx.gmm_last_path() == fg.GMM_PATH_FP32
+    assert abs(Nk.sum() - N) <= 1e-5 * N
+    np.testing.assert_allclose(S2.sum(0), col2, rtol=1e-4)
+    np.testing.assert_allclose(S1.sum(0), col1, rtol=1e-4, atol=1e-4 * N * 0.04)
+    # parameters after one update (sharper responsibilities) for the top-m check
+    pi_d, mu_d, var_d = _t(pi0), _t(mu0), _t(var0)
+    ctx.gmm_finalize(N, _t(Nk, torch.float64), _t(S1, torch.float64), _t(S2, torch.float64), spec.var_floor, pi_d, mu_d,
+                     var_d)
+    idx, resp = ctx.gmm_assign_topm(X, pi_d, mu_d, var_d, 4)
+    torch.cuda.synchronize()
+    rows = synth.subsample_rows(N, 20_000, spec.seed)
+    rows_d = torch.as_tensor(rows, device=DEV)
+    Xsub_d = X[rows_d].contiguous()
+    Xsub = Xsub_d.cpu().numpy()
+    ref = orc.em_step(Xsub, pi0, mu0, var0)
+    got = _gpu_step(ctx, Xsub_d, pi0, mu0, var0)
+    assert abs(got[3] - ref[3]) <= 1e-5 * abs(ref[3])
+    assert_stats_close(len(rows), data_scale(Xsub), got[:3], ref[:3], "config 5 subsample")
+    p1, m1, v1 = pi_d.cpu().numpy(), mu_d.cpu().numpy(), var_d.cpu().numpy()
+    idx_r, resp_r, next_r = orc.topm(Xsub, p1, m1, v1, 4)
+    assert_topm_matches(idx[rows_d].cpu().numpy(), resp[rows_d].cpu().numpy(), idx_r, resp_r, next_r,
+                        what="config 5 top-4 subsample")

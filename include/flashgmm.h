@@ -48,6 +48,10 @@ extern "C" {
 #define GMM_PATH_FP32   1  /* CUDA-core float32 kernels with direct differences (x - mu)^2 / var; any shape */
 #define GMM_PATH_TENSOR 2  /* tcgen05 tensor-core kernels on the expanded quadratic form; restricted shapes */
 
+/* Covariance model used by the parameter update of gmm_fit (gmm_set_covariance). */
+#define GMM_COV_DIAG      0  /* per-dimension variances (default) */
+#define GMM_COV_ISOTROPIC 1  /* the paper's sigma_k^2 I: one variance per component, stored replicated over d */
+
 #define GMM_MAX_TOPM 8
 
 typedef struct gmm_ctx gmm_ctx;
@@ -98,6 +102,16 @@ int gmm_em_step_host(gmm_ctx* ctx, const float* X_host, int64_t N, int D, int K,
 int gmm_finalize(gmm_ctx* ctx, int64_t N, int D, int K,
                  const double* Nk, const double* S1, const double* S2,
                  float var_floor, float* pi, float* mu, float* var);
+
+/* The paper's own update (Section 2, Eq. 3; Algorithm 1's last line) for the isotropic model sigma_k^2 I:
+ *   sigma_k^2 = (1 / (D N_k)) sum_i r_ik ||x_i - mu_k^new||^2 = (1 / (D N_k)) sum_d (S2_kd - N_k mu_kd^2),
+ * floored at var_floor and written to all D entries of var[k, :], so that gmm_em_step / gmm_assign_topm evaluate
+ * N(x | mu_k, sigma_k^2 I) with the same kernels.  Same arguments and rules as gmm_finalize. */
+int gmm_finalize_isotropic(gmm_ctx* ctx, int64_t N, int D, int K,
+                           const double* Nk, const double* S1, const double* S2,
+                           float var_floor, float* pi, float* mu, float* var);
+/* Selects which update gmm_fit applies: GMM_COV_DIAG (default) or GMM_COV_ISOTROPIC. */
+int gmm_set_covariance(gmm_ctx* ctx, int covariance);
 
 /* EM driver: `iters` iterations of gmm_em_step + gmm_finalize (paper Section 2, last paragraph; Algorithm 1 run
  * repeatedly).  pi/mu/var: device, in = initial parameters, out = fitted.  loglik_trace: host [iters];

@@ -277,6 +277,64 @@ int oracle_em_iteration(const float* X, int64_t N, int D, int K, double* pi, dou
     return 0;
 }
 
+// The paper's own model: isotropic covariance sigma_k^2 I.  One EM iteration exactly as Section 2 states it: E-step,
+// Eq. 1, pi_k = N_k / N, Eq. 2, and Eq. 3  sigma_k^2 = (1 / (D N_k)) sum_i r_ik ||x_i - mu_k^new||^2  (new mean; second pass
+// with the responsibilities recomputed from the OLD parameters).  var holds one value per component replicated over d
+// (so the same E-step code evaluates N(x | mu_k, sigma_k^2 I)); it is in (old) / out (new).
+int oracle_em_iteration_isotropic(const float* X, int64_t N, int D, int K, double* pi, double* mu, double* var,
+                                  double var_floor, double* loglik, int nthreads) {
+    if (!X || !pi || !mu || !var || !loglik || N < 1 || D < 1 || K < 1) return -1;
+    const size_t KD = (size_t)K * D;
+    std::vector<double> Nk(K), S1(KD), S2(KD);
+    int rc = oracle_em_step(X, N, D, K, pi, mu, var, Nk.data(), S1.data(), S2.data(), loglik, nthreads);
+    if (rc) return rc;
+    std::vector<double> mu_new(mu, mu + KD);
+    for (int k = 0; k < K; ++k) {
+        if (Nk[k] < 1e-12) continue;
+        for (int d = 0; d < D; ++d) mu_new[(size_t)k * D + d] = S1[(size_t)k * D + d] / Nk[k];      // Eq. 2
+    }
+    const int T = clamp_threads(nthreads);
+    const Prepared pre(D, K, pi, var);
+    std::vector<std::vector<double>> pQ(T);
+#pragma omp parallel num_threads(T)
+    {
+#ifdef _OPENMP
+        const int t = omp_get_thread_num();
+#else
+        const int t = 0;
+#endif
+        pQ[t].assign(K, 0.0);
+        std::vector<double> ell(K), r(K);
+        const int64_t lo = N * t / T, hi = N * (t + 1) / T;
+        for (int64_t i = lo; i < hi; ++i) {
+            const float* x = X + i * D;
+            point_responsibilities(x, D, K, pre, mu, ell.data(), r.data());
+            for (int k = 0; k < K; ++k) {
+                if (r[k] == 0.0) continue;
+                const double* m = mu_new.data() + (size_t)k * D;
+                double sq = 0.0;
+                for (int d = 0; d < D; ++d) {
+                    const double diff = (double)x[d] - m[d];
+                    sq += diff * diff;
+                }
+                pQ[t][k] += r[k] * sq;                                                              // r_ik ||x_i - mu_k||^2
+            }
+        }
+    }
+    for (int k = 0; k < K; ++k) {
+        pi[k] = Nk[k] / (double)N;
+        if (Nk[k] < 1e-12) continue;
+        double Q = 0.0;
+        for (int t = 0; t < T; ++t) Q += pQ[t][k];
+        const double v = std::max(Q / ((double)D * Nk[k]), var_floor);                              // Eq. 3
+        for (int d = 0; d < D; ++d) {
+            mu[(size_t)k * D + d] = mu_new[(size_t)k * D + d];
+            var[(size_t)k * D + d] = v;
+        }
+    }
+    return 0;
+}
+
 // EM driver: iters iterations from the given parameters (in/out).  trace[t] = log-likelihood under the
 // parameters ENTERING iteration t.  If params_trace is non-null it receives the parameters entering each
 // iteration, laid out [iters+1][K + 2*K*D] as (pi, mu, var), the last block being the final parameters.

@@ -68,6 +68,7 @@ def _load():
         "oracle_em_step": ([c_fp, i64, ci, ci, c_dp, c_dp, c_dp, c_dp, c_dp, c_dp, c_dp, ci], ci),
         "oracle_finalize_moments": ([i64, ci, ci, c_dp, c_dp, c_dp, ctypes.c_double, c_dp, c_dp, c_dp], ci),
         "oracle_em_iteration": ([c_fp, i64, ci, ci, c_dp, c_dp, c_dp, ctypes.c_double, c_dp, c_dp, c_dp, ci], ci),
+        "oracle_em_iteration_isotropic": ([c_fp, i64, ci, ci, c_dp, c_dp, c_dp, ctypes.c_double, c_dp, ci], ci),
         "oracle_fit": ([c_fp, i64, ci, ci, c_dp, c_dp, c_dp, ci, ctypes.c_double, ctypes.c_double, c_dp,
                         ctypes.POINTER(ci), c_dp, ci], ci),
         "oracle_topm": ([c_fp, i64, ci, ci, c_dp, c_dp, c_dp, ci, c_ip, c_dp, c_dp, ci], ci),
@@ -189,6 +190,19 @@ def em_iteration(X, pi, mu, var, var_floor: float = 0.0, nthreads: int = 0):
                                      _dp(Nk), _dp(S1), nthreads)
     _check(rc, "oracle_em_iteration")
     return pi, mu, var, L.value, Nk, S1
+
+
+def em_iteration_isotropic(X, pi, mu, var, var_floor: float = 0.0, nthreads: int = 0):
+    """One EM iteration of the paper's isotropic model (Eq. 1-3 as printed).  ``var`` is [K, D] with each row constant.
+
+    Returns (pi_new, mu_new, var_new [K, D] with constant rows, loglik_under_old_params)."""
+    X, mu, N, D, K = _shapes(X, mu)
+    pi, mu, var = _f64(pi).copy(), mu.copy(), _f64(var).copy()
+    L = ctypes.c_double(0.0)
+    rc = _load().oracle_em_iteration_isotropic(_fp(X), N, D, K, _dp(pi), _dp(mu), _dp(var), float(var_floor),
+                                               ctypes.byref(L), nthreads)
+    _check(rc, "oracle_em_iteration_isotropic")
+    return pi, mu, var, L.value
 
 
 def fit(X, pi, mu, var, iters: int, var_floor: float = 0.0, tol: float = 0.0, keep_params: bool = False,

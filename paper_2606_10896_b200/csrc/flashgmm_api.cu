@@ -75,6 +75,7 @@ struct gmm_ctx {
     cudaStream_t stream = nullptr;
     int path = GMM_PATH_AUTO;
     int last_path = 0;
+    int covariance = GMM_COV_DIAG;
     // scratch
     unsigned char* scratch = nullptr;
     size_t scratch_bytes = 0;
@@ -416,6 +417,28 @@ int gmm_finalize(gmm_ctx* ctx, int64_t N, int D, int K, const double* Nk, const 
     return GMM_OK;
 }
 
+int gmm_set_covariance(gmm_ctx* ctx, int covariance) {
+    if (!ctx) return GMM_EINVAL;
+    if (covariance != GMM_COV_DIAG && covariance != GMM_COV_ISOTROPIC) return fail(ctx, GMM_EINVAL, "unknown covariance type %d", covariance);
+    ctx->covariance = covariance;
+    return GMM_OK;
+}
+
+int gmm_finalize_isotropic(gmm_ctx* ctx, int64_t N, int D, int K, const double* Nk, const double* S1, const double* S2,
+                           float var_floor, float* pi, float* mu, float* var) {
+    CHECK(check_shape(ctx, N, D, K));
+    CHECK(check_ptr(ctx, Nk, 8, "Nk"));
+    CHECK(check_ptr(ctx, S1, 8, "S1"));
+    CHECK(check_ptr(ctx, S2, 8, "S2"));
+    CHECK(check_ptr(ctx, pi, 4, "pi"));
+    CHECK(check_ptr(ctx, mu, 4, "mu"));
+    CHECK(check_ptr(ctx, var, 4, "var"));
+    if (!(var_floor >= 0.f)) return fail(ctx, GMM_EINVAL, "var_floor must be >= 0");
+    DeviceGuard g(ctx->device);
+    KL(launch_finalize_isotropic(ctx->stream, N, D, K, Nk, S1, S2, var_floor, pi, mu, var));
+    return GMM_OK;
+}
+
 int gmm_fit(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, float* pi, float* mu, float* var, int iters,
             float var_floor, double tol, double* loglik_trace, int* iters_done) {
     CHECK(check_shape(ctx, N, D, K));
@@ -440,7 +463,10 @@ int gmm_fit(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, float* pi, fl
         CHECK(prepare_and_choose(ctx, N, D, K, pi, mu, var, &path));
         CHECK(zero_stats(ctx, D, K, Nk, S1, S2, slot));
         CHECK(accumulate_points(ctx, path, X, N, D, K, mu, Nk, S1, S2, slot));
-        KL(launch_finalize(ctx->stream, N, D, K, Nk, S1, S2, var_floor, pi, mu, var));
+        if (ctx->covariance == GMM_COV_ISOTROPIC)
+            KL(launch_finalize_isotropic(ctx->stream, N, D, K, Nk, S1, S2, var_floor, pi, mu, var));
+        else
+            KL(launch_finalize(ctx->stream, N, D, K, Nk, S1, S2, var_floor, pi, mu, var));
         ctx->last_path = path;
         int rc = read_result(ctx, slot, &loglik_trace[t]);
         if (rc != GMM_OK) {

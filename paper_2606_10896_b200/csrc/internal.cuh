@@ -48,4 +48,7 @@ cudaError_t launch_reduce_ll(cudaStream_t s, const double* llpart, int64_t n, do
 cudaError_t launch_finalize(cudaStream_t s, int64_t N, int D, int K, const double* Nk, const double* S1,
                             const double* S2, float var_floor, float* pi, float* mu, float* var);
 
+cudaError_t launch_finalize_isotropic(cudaStream_t s, int64_t N, int D, int K, const double* Nk, const double* S1,
+                                      const double* S2, float var_floor, float* pi, float* mu, float* var);
+
 }  // namespace fg

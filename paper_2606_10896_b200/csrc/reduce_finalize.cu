@@ -51,7 +51,43 @@ __global__ void finalize_kernel(int64_t N, int D, int K, const double* __restric
     var[e] = (float)v;
 }
 
+// The paper's isotropic model: sigma_k^2 = (1 / (D N_k)) sum_i r_ik ||x_i - mu_k^new||^2 (Eq. 3), which in terms of the
+// statistics is (1 / (D N_k)) sum_d (S2_kd - N_k mu_kd^2).  One block per component; the value is written to all D
+// entries of var so that every other entry point sees an ordinary diagonal model.
+__global__ void finalize_isotropic_kernel(int64_t N, int D, int K, const double* __restrict__ Nk,
+                                          const double* __restrict__ S1, const double* __restrict__ S2,
+                                          float var_floor, float* __restrict__ pi, float* __restrict__ mu,
+                                          float* __restrict__ var) {
+    const int k = blockIdx.x;
+    __shared__ double red[128];
+    const double nk = Nk[k];
+    if (threadIdx.x == 0) pi[k] = (float)(nk / (double)N);
+    if (nk < 1e-12) return;
+    double q = 0.0;
+    for (int d = threadIdx.x; d < D; d += blockDim.x) {
+        const double m = S1[(size_t)k * D + d] / nk;
+        q += S2[(size_t)k * D + d] - nk * m * m;
+        mu[(size_t)k * D + d] = (float)m;
+    }
+    red[threadIdx.x] = q;
+    __syncthreads();
+    for (int o = blockDim.x / 2; o > 0; o >>= 1) {
+        if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o];
+        __syncthreads();
+    }
+    double v = red[0] / ((double)D * nk);
+    const double fl = (double)var_floor;
+    if (!(v > fl)) v = fl;
+    for (int d = threadIdx.x; d < D; d += blockDim.x) var[(size_t)k * D + d] = (float)v;
+}
+
 }  // namespace
+
+cudaError_t launch_finalize_isotropic(cudaStream_t s, int64_t N, int D, int K, const double* Nk, const double* S1,
+                                      const double* S2, float var_floor, float* pi, float* mu, float* var) {
+    finalize_isotropic_kernel<<<K, 128, 0, s>>>(N, D, K, Nk, S1, S2, var_floor, pi, mu, var);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_reduce_partials(cudaStream_t s, int D, int K, int splits, const float* partials, double* Nk,
                                    double* S1, double* S2, bool accumulate) {

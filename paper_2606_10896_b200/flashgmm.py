@@ -19,6 +19,7 @@ GMM_OK = 0
 GMM_EINVAL, GMM_EALIGN, GMM_ENOMEM, GMM_ECUDA, GMM_ENUMERIC, GMM_ETIMEOUT, GMM_EUNSUPPORTED = -1, -2, -3, -4, -5, -6, -7
 GMM_PATH_AUTO, GMM_PATH_FP32, GMM_PATH_TENSOR = 0, 1, 2
 GMM_MAX_TOPM = 8
+GMM_COV_DIAG, GMM_COV_ISOTROPIC = 0, 1
 
 EXPORTS = {
     # name: (restype, argtypes)
@@ -39,6 +40,10 @@ EXPORTS = {
     "gmm_finalize": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_int,
                                     ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_float,
                                     ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
+    "gmm_finalize_isotropic": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_int,
+                                              ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_float,
+                                              ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
+    "gmm_set_covariance": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int]),
     "gmm_fit": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_int,
                                ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                ctypes.c_int, ctypes.c_float, ctypes.c_double,
@@ -235,6 +240,18 @@ class Context:
                               float(var_floor), _dev(pi, torch.float32, (K,), "pi"),
                               _dev(mu, torch.float32, (K, D), "mu"), _dev(var, torch.float32, (K, D), "var"))
         self._check(rc)
+
+    def gmm_finalize_isotropic(self, N, Nk, S1, S2, var_floor, pi, mu, var):
+        """In-place update for the paper's isotropic model (one variance per component, replicated over d)."""
+        K, D = mu.shape
+        rc = lib.gmm_finalize_isotropic(self._h, int(N), D, K, _dev(Nk, torch.float64, (K,), "Nk"),
+                                        _dev(S1, torch.float64, (K, D), "S1"), _dev(S2, torch.float64, (K, D), "S2"),
+                                        float(var_floor), _dev(pi, torch.float32, (K,), "pi"),
+                                        _dev(mu, torch.float32, (K, D), "mu"), _dev(var, torch.float32, (K, D), "var"))
+        self._check(rc)
+
+    def gmm_set_covariance(self, covariance: int):
+        self._check(lib.gmm_set_covariance(self._h, int(covariance)))
 
     def gmm_fit(self, X, pi, mu, var, iters, var_floor=1e-6, tol=0.0):
         """Runs EM in place on pi, mu, var; returns (loglik_trace float64 numpy [iters_done], iters_done)."""

@@ -333,3 +333,25 @@ def test_topm_ties_go_to_smaller_index():
     idx, resp, _ = orc.topm(X, np.full(4, 0.25), mu, np.ones((4, 2)), 2)
     np.testing.assert_array_equal(idx, [[0, 1]] * 3)
     np.testing.assert_allclose(resp, 0.25)
+
+
+def test_isotropic_iteration_is_eq3_as_printed():
+    """The isotropic oracle against the paper's Eq. 1-3 evaluated from library responsibilities, and against the mean
+    over d of the diagonal update (the two must coincide when the old variances are isotropic)."""
+    X, pi, mu, _ = _random_problem(21, 500, 5, 4)
+    s2 = np.array([0.8, 1.4, 0.5, 2.0])
+    var = np.repeat(s2[:, None], 5, axis=1)
+    Xd = X.astype(np.float64)
+    Rl, lzl = _library_responsibilities(X, pi, mu, var)
+    pn, mn, vn, L = orc.em_iteration_isotropic(X, pi, mu, var)
+    assert L == pytest.approx(lzl.sum(), rel=1e-13)
+    for k in range(4):
+        Nk = Rl[:, k].sum()
+        m = (Rl[:, k, None] * Xd).sum(0) / Nk                                   # Eq. 2
+        v = (Rl[:, k] * ((Xd - m) ** 2).sum(1)).sum() / (5 * Nk)                # Eq. 3
+        assert pn[k] == pytest.approx(Nk / len(X), rel=1e-11)
+        np.testing.assert_allclose(mn[k], m, rtol=1e-10, atol=1e-12)
+        np.testing.assert_allclose(vn[k], v, rtol=1e-10)                        # every d carries the same value
+    _, md, vd, _, _, _ = orc.em_iteration(X, pi, mu, var)
+    np.testing.assert_allclose(mn, md, rtol=1e-13)
+    np.testing.assert_allclose(vn[:, 0], vd.mean(1), rtol=1e-10)

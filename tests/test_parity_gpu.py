@@ -428,3 +428,37 @@ def test_config5_shape_step_and_topm_on_subsample(fg, ctx):
     idx_r, resp_r, next_r = orc.topm(Xsub, p1, m1, v1, 4)
     assert_topm_matches(idx[rows_d].cpu().numpy(), resp[rows_d].cpu().numpy(), idx_r, resp_r, next_r,
                         what="config 5 top-4 subsample")
+
+
+def test_isotropic_update_and_fit_match_the_papers_model(fg, ctx):
+    """gmm_finalize_isotropic and gmm_fit with GMM_COV_ISOTROPIC against the isotropic oracle (the paper's Eq. 3)."""
+    spec = synth.CONFIGS[2].with_n(6000)
+    X = synth.sample_host(spec)
+    s = data_scale(X)
+    pi0, mu0, var0 = synth.init_params(X, spec)
+    var0 = np.full_like(var0, var0.mean())                       # isotropic start: sigma^2 = mean global variance
+    pr, mr, vr, L_r = orc.em_iteration_isotropic(X, pi0, mu0, var0, spec.var_floor)
+    Nk_r = orc.em_step(X, pi0, mu0, var0)[0]
+    for path in _paths(fg, spec.D, spec.K):
+        ctx.gmm_set_path(path)
+        Nk, S1, S2, L = ctx.gmm_em_step(_t(X), _t(pi0), _t(mu0), _t(var0))
+        assert abs(L - L_r) <= 1e-5 * abs(L_r)
+        pi_d, mu_d, var_d = _t(pi0), _t(mu0), _t(var0)
+        ctx.gmm_finalize_isotropic(len(X), Nk, S1, S2, spec.var_floor, pi_d, mu_d, var_d)
+        v = var_d.cpu().numpy()
+        assert (v == v[:, :1]).all()
+        assert_params_close(len(X), s, (pi_d.cpu().numpy(), mu_d.cpu().numpy(), v), (pr, mr, vr), Nk_r, f"path {path}")
+    # gmm_fit with the isotropic update, teacher-forced: one iteration at a time from the oracle's parameters
+    ctx.gmm_set_path(fg.GMM_PATH_AUTO)
+    ctx.gmm_set_covariance(fg.GMM_COV_ISOTROPIC)
+    p, m, v = pi0.astype(np.float64), mu0.astype(np.float64), var0.astype(np.float64)
+    for it in range(3):
+        p32, m32, v32 = p.astype(np.float32), m.astype(np.float32), v.astype(np.float32)
+        Nk_it = orc.em_step(X, p32, m32, v32)[0]
+        p, m, v, L = orc.em_iteration_isotropic(X, p32, m32, v32, spec.var_floor)
+        pi_d, mu_d, var_d = _t(p32), _t(m32), _t(v32)
+        trace, done = ctx.gmm_fit(_t(X), pi_d, mu_d, var_d, 1, spec.var_floor)
+        assert done == 1 and abs(trace[0] - L) <= 1e-5 * abs(L)
+        assert_params_close(len(X), s, (pi_d.cpu().numpy(), mu_d.cpu().numpy(), var_d.cpu().numpy()), (p, m, v), Nk_it,
+                            f"isotropic fit iteration {it}")
+    ctx.gmm_set_covariance(fg.GMM_COV_DIAG)

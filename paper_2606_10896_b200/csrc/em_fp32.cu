@@ -347,6 +347,127 @@ mstep_kernel(const float* __restrict__ X, int64_t n, int D, int K, const float* 
     }
 }
 
+// M-step for D > 128.  A CTA owns 64 components and ALL of D: it forms the responsibilities of a batch of WT point
+// tiles once (full-D quadratic forms, float64 logits) and keeps them in shared memory, then sweeps the 128-wide slices
+// of D, accumulating each slice over the whole batch in registers and adding it to this CTA's own rows of a float64
+// partial in global memory (no other CTA touches them: deterministic, no atomics).  The E-step is thus recomputed once
+// per point and component, not once per slice of D.
+constexpr int WT = 6;
+constexpr size_t MSTEP_WIDE_SMEM = sizeof(TileSmem) + (size_t)WT * TP * LDR * 4 + (size_t)TP * LDX * 4;
+
+__global__ void __launch_bounds__(NTHREADS)
+mstep_wide_kernel(const float* __restrict__ X, int64_t n, int D, int K, const float* __restrict__ mu,
+                  const float* __restrict__ w2, const double* __restrict__ c2, const double* __restrict__ logZ2,
+                  double* __restrict__ partials) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    TileSmem& sm = *reinterpret_cast<TileSmem*>(smem_raw);
+    float* r_all = reinterpret_cast<float*>(smem_raw + sizeof(TileSmem));   // [WT][TP][LDR]
+    float* xm = r_all + WT * TP * LDR;                                       // [TP][LDX]
+    const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+    const int kq = tid >> 5, dq = tid & 31;
+    const int k0 = blockIdx.x * TC;
+    const int split = blockIdx.y, nsplits = gridDim.y;
+    const int64_t ntiles = (n + TP - 1) / TP;
+    const int d_chunks = (D + FP32_MSTEP_DC - 1) / FP32_MSTEP_DC;
+    const size_t KD = (size_t)K * D;
+    double* pN = partials + (size_t)split * (K + 2 * KD);
+    double* pS1 = pN + K;
+    double* pS2 = pS1 + KD;
+
+    double cv[4];
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+        const int k = k0 + 4 * tx + b;
+        cv[b] = (k < K) ? __ldg(c2 + k) : (double)(-CUDART_INF_F);
+    }
+    double nacc = 0.0;
+
+    for (int64_t t0 = split; t0 < ntiles; t0 += (int64_t)nsplits * WT) {
+        // ---- responsibilities of the batch (tiles t0, t0 + nsplits, ...) ----
+        int nb = 0;
+        for (int w = 0; w < WT; ++w) {
+            const int64_t t = t0 + (int64_t)w * nsplits;
+            if (t >= ntiles) break;
+            ++nb;
+            const int64_t row0 = t * TP;
+            double q[4][4];
+            tile_quadratic<double>(sm, X, row0, n, D, mu, w2, k0, K, q);
+            float* r_s = r_all + w * TP * LDR;
+#pragma unroll
+            for (int a = 0; a < 4; ++a) {
+                const int64_t row = row0 + 4 * ty + a;
+                const double lz = (row < n) ? __ldg(logZ2 + row) : (double)CUDART_INF_F;
+                float4 rv;
+                rv.x = fast_ex2((float)(cv[0] - q[a][0] - lz));
+                rv.y = fast_ex2((float)(cv[1] - q[a][1] - lz));
+                rv.z = fast_ex2((float)(cv[2] - q[a][2] - lz));
+                rv.w = fast_ex2((float)(cv[3] - q[a][3] - lz));
+                *reinterpret_cast<float4*>(&r_s[(4 * ty + a) * LDR + 4 * tx]) = rv;
+            }
+        }
+        __syncthreads();
+        if (tid < TC) {
+            float s = 0.f;
+            for (int w = 0; w < nb; ++w)
+                for (int i = 0; i < TP; ++i) s += r_all[(w * TP + i) * LDR + tid];
+            nacc += (double)s;
+        }
+        // ---- sweep the slices of D ----
+        for (int dz = 0; dz < d_chunks; ++dz) {
+            const int dz0 = dz * FP32_MSTEP_DC;
+            float acc1[8][4], acc2[8][4];
+#pragma unroll
+            for (int c = 0; c < 8; ++c)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) { acc1[c][j] = 0.f; acc2[c][j] = 0.f; }
+            for (int w = 0; w < nb; ++w) {
+                const int64_t row0 = (t0 + (int64_t)w * nsplits) * TP;
+                __syncthreads();
+#pragma unroll 4
+                for (int j = 0; j < (TP * FP32_MSTEP_DC) / NTHREADS; ++j) {
+                    const int e = tid + j * NTHREADS, r = e >> 7, c = e & 127;
+                    const int64_t row = row0 + r;
+                    const int d = dz0 + c;
+                    xm[r * LDX + c] = (row < n && d < D) ? __ldg(X + row * D + d) : 0.f;
+                }
+                __syncthreads();
+                const float* r_s = r_all + w * TP * LDR;
+#pragma unroll 2
+                for (int i = 0; i < TP; ++i) {
+                    const float4 xv = *reinterpret_cast<const float4*>(&xm[i * LDX + 4 * dq]);
+                    const float4 ra = *reinterpret_cast<const float4*>(&r_s[i * LDR + 8 * kq]);
+                    const float4 rb = *reinterpret_cast<const float4*>(&r_s[i * LDR + 8 * kq + 4]);
+                    const float x1[4] = {xv.x, xv.y, xv.z, xv.w};
+                    const float x2[4] = {xv.x * xv.x, xv.y * xv.y, xv.z * xv.z, xv.w * xv.w};
+                    const float rr[8] = {ra.x, ra.y, ra.z, ra.w, rb.x, rb.y, rb.z, rb.w};
+#pragma unroll
+                    for (int c = 0; c < 8; ++c)
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            acc1[c][j] = fmaf(rr[c], x1[j], acc1[c][j]);
+                            acc2[c][j] = fmaf(rr[c], x2[j], acc2[c][j]);
+                        }
+                }
+            }
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                const int k = k0 + 8 * kq + c;
+                if (k >= K) continue;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int d = dz0 + 4 * dq + j;
+                    if (d < D) {
+                        pS1[(size_t)k * D + d] += (double)acc1[c][j];
+                        pS2[(size_t)k * D + d] += (double)acc2[c][j];
+                    }
+                }
+            }
+        }
+        __syncthreads();      // r_all is rewritten by the next batch
+    }
+    if (tid < TC && k0 + tid < K) pN[k0 + tid] = nacc;
+}
+
 // One block per component: w2 = (log2 e / 2) / var, c2 = log2 e (log pi - 1/2 sum_d log(2 pi var)), in float64.
 __global__ void prepare_fp32_kernel(int D, int K, const float* __restrict__ pi, const float* __restrict__ mu,
                                     const float* __restrict__ var, float* __restrict__ w2, float* __restrict__ c2,
@@ -387,15 +508,19 @@ Fp32Plan fp32_plan(int D, int K) {
     Fp32Plan p;
     p.comp_blocks = (K + TC - 1) / TC;
     p.d_chunks = (D + FP32_MSTEP_DC - 1) / FP32_MSTEP_DC;
-    const int per = p.comp_blocks * p.d_chunks;
-    p.splits = (FP32_TARGET_CTAS + per - 1) / per;
+    p.wide = D > FP32_MSTEP_DC;
+    // wide shapes: one CTA loops over the D slices itself (one resident CTA per SM: float64 logits are register-hungry)
+    const int per = p.wide ? p.comp_blocks : p.comp_blocks * p.d_chunks;
+    const int target = p.wide ? 148 : FP32_TARGET_CTAS;
+    p.splits = (target + per - 1) / per;
     if (p.splits < 1) p.splits = 1;
     return p;
 }
 
 size_t fp32_partial_floats(int D, int K) {
     const Fp32Plan p = fp32_plan(D, K);
-    return (size_t)p.splits * ((size_t)K + 2 * (size_t)K * D);
+    // wide shapes keep float64 partials (they are accumulated into across batches of tiles)
+    return (size_t)p.splits * ((size_t)K + 2 * (size_t)K * D) * (p.wide ? 2 : 1);
 }
 
 cudaError_t launch_prepare_fp32(cudaStream_t s, int D, int K, const float* pi, const float* mu, const float* var,
@@ -447,6 +572,16 @@ cudaError_t launch_topm_fp32(cudaStream_t s, const float* X, int64_t n, int D, i
 cudaError_t launch_mstep_fp32(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu,
                               const float* w2, const double* c2d, const double* logZ2, float* partials,
                               const Fp32Plan& plan) {
+    if (plan.wide) {
+        cudaError_t e = cudaFuncSetAttribute(mstep_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)MSTEP_WIDE_SMEM);
+        if (e != cudaSuccess) return e;
+        const size_t bytes = (size_t)plan.splits * ((size_t)K + 2 * (size_t)K * D) * sizeof(double);
+        e = cudaMemsetAsync(partials, 0, bytes, s);          // the kernel accumulates into its partials
+        if (e != cudaSuccess) return e;
+        dim3 wgrid(plan.comp_blocks, plan.splits, 1);
+        mstep_wide_kernel<<<wgrid, NTHREADS, MSTEP_WIDE_SMEM, s>>>(X, n, D, K, mu, w2, c2d, logZ2, reinterpret_cast<double*>(partials));
+        return cudaGetLastError();
+    }
     dim3 grid(plan.comp_blocks, plan.splits, plan.d_chunks);
     if (fp32_high_precision(D)) {
         cudaError_t e = cudaFuncSetAttribute(mstep_kernel<double>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)MSTEP_SMEM);

@@ -41,7 +41,8 @@ StaticLayout static_layout(int D, int K) {
     StaticLayout L;
     const size_t KD = (size_t)K * D;
     Fp32Plan plan = fp32_plan(D, K);
-    L.splits = plan.splits < STATIC_MAX_SPLITS ? plan.splits : STATIC_MAX_SPLITS;
+    const int max_splits = plan.wide ? STATIC_MAX_SPLITS / 2 : STATIC_MAX_SPLITS;   // float64 partials when wide
+    L.splits = plan.splits < max_splits ? plan.splits : max_splits;
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off += al(bytes); return o; };
     L.w2 = take(KD * 4);
@@ -50,7 +51,7 @@ StaticLayout static_layout(int D, int K) {
     L.logZ2 = take((size_t)STATIC_TILE * 8);
     L.llpart = take((size_t)(STATIC_TILE / FP32_TILE_P) * 8);
     L.result = take(sizeof(StaticResult));
-    L.partials = take((size_t)L.splits * ((size_t)K + 2 * KD) * 4);
+    L.partials = take((size_t)L.splits * ((size_t)K + 2 * KD) * (plan.wide ? 8 : 4));
     L.total = off;
     return L;
 }

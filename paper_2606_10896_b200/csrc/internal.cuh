@@ -21,6 +21,7 @@ enum : int { ST_BAD_VAR = 1, ST_BAD_PI = 2, ST_NONFINITE = 4, ST_TIMEOUT = 8, ST
 
 struct Fp32Plan {
     int comp_blocks, d_chunks, splits;
+    bool wide;      // D > 128: one CTA sweeps all slices of D; partials are float64
 };
 Fp32Plan fp32_plan(int D, int K);
 size_t fp32_partial_floats(int D, int K);   // floats in the per-CTA partial buffer
@@ -40,7 +41,7 @@ cudaError_t launch_topm_fp32(cudaStream_t s, const float* X, int64_t n, int D, i
 
 // ---- shared by all paths -------------------------------------------------------------------------------------
 // stats (+)= sum over `splits` partial blocks, fixed order, float64.  Partial layout: [splits][K + 2*K*D] floats,
-// each block being (N_k [K], S1 [K*D], S2 [K*D]).
+// each block being (N_k [K], S1 [K*D], S2 [K*D]); float64 instead when fp32_plan(D, K).wide.
 cudaError_t launch_reduce_partials(cudaStream_t s, int D, int K, int splits, const float* partials, double* Nk,
                                    double* S1, double* S2, bool accumulate);
 // *ll (+)= sum of llpart[0..n) in a fixed order

@@ -7,7 +7,8 @@ namespace fg {
 
 namespace {
 
-__global__ void reduce_partials_kernel(int D, int K, int splits, const float* __restrict__ partials,
+template <typename T>
+__global__ void reduce_partials_kernel(int D, int K, int splits, const T* __restrict__ partials,
                                        double* __restrict__ Nk, double* __restrict__ S1, double* __restrict__ S2,
                                        int accumulate) {
     const size_t KD = (size_t)K * D, per = (size_t)K + 2 * KD;
@@ -93,7 +94,11 @@ cudaError_t launch_reduce_partials(cudaStream_t s, int D, int K, int splits, con
                                    double* S1, double* S2, bool accumulate) {
     const size_t per = (size_t)K + 2 * (size_t)K * D;
     const unsigned blocks = (unsigned)((per + 255) / 256);
-    reduce_partials_kernel<<<blocks, 256, 0, s>>>(D, K, splits, partials, Nk, S1, S2, accumulate ? 1 : 0);
+    if (fp32_plan(D, K).wide)
+        reduce_partials_kernel<double><<<blocks, 256, 0, s>>>(D, K, splits, reinterpret_cast<const double*>(partials), Nk, S1, S2,
+                                                              accumulate ? 1 : 0);
+    else
+        reduce_partials_kernel<float><<<blocks, 256, 0, s>>>(D, K, splits, partials, Nk, S1, S2, accumulate ? 1 : 0);
     return cudaGetLastError();
 }
 

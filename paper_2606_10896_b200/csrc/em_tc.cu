@@ -26,6 +26,9 @@
 #include "em_tc.cuh"
 
 #include <cuda_fp16.h>
+#ifdef FLASHGMM_DEBUG
+#include <cstdio>
+#endif
 #include <math_constants.h>
 
 namespace fg {
@@ -120,6 +123,12 @@ __device__ __forceinline__ void mma_commit(uint32_t bar) {
 __device__ __forceinline__ void fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// One lane of a converged warp (all 32 lanes must call it together).
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xffffffff;\n\tselp.u32 %0, 1, 0, P;\n\t}\n" : "=r"(pred)::"memory");
+    return pred != 0u;
+}
 
 __device__ __forceinline__ void bar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
@@ -313,6 +322,8 @@ struct TcKernelParams {
     int* status;
 #ifdef FLASHGMM_DEBUG
     float* dbg;      // [Kpad][64] log2 z of the first tile
+    int dbg_cluster, dbg_i; // which (group, local tile) the logit dump records
+    uint4* dbg_y;           // [4096] copy of the Y stage as the issuer finds it after its wait (CTA rank 0 of the group)
     long long* dbg_clk;   // per-phase cycle counters of CTA 0
     long long* dbg_trace; // [64 tiles][16 events] clock64 stamps of CTA 0
 #endif
@@ -439,7 +450,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                 for (int j = 0; j < 32; ++j) l[j] = fmaf(__uint_as_float(v0[j]), tk, ck);
             }
 #ifdef FLASHGMM_DEBUG
-            if (p.dbg && cluster_id == 0 && i == 0)
+            if (p.dbg && cluster_id == p.dbg_cluster && i == p.dbg_i)
                 for (int j = 0; j < 32; ++j) p.dbg[(size_t)(rank * 128 + kloc) * 64 + p0 + j] = l[j];
 #endif
             TOC(tk_, 16);
@@ -739,34 +750,59 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
             TOC(tt_, 11);
             if (tau == 0) TRACE(6, i);
         }
-    } else if (lane == 0) {
-        // =========================== MMA issuer (one thread) ===========================
+    } else {
+        // =========================== MMA warp ===========================
+        // The whole warp runs this loop convergently; lane 0 does the (bounded) waits and broadcasts their outcome, one
+        // elected lane issues the MMAs and commits, and the warp meets again after every batch.
         const uint32_t id_e = make_idesc(128, BN, 0);
         const uint32_t id_m = make_idesc(128, p.n_ks * 16, 1);
-        const uint32_t plo = smem_u32(smem + SM_PLO);
+        const int n_ks = p.n_ks;
+        // Descriptors are hoisted bases plus compile-time offsets (address field, 16-byte units): the issuing thread must
+        // spend only a few instructions per MMA or it, not the tensor pipe, sets the pace.
+        const uint64_t d_plo = make_desc(smem_u32(smem + SM_PLO), 16, 1024);
+        const uint32_t y0 = smem_u32(smem + SM_Y);
         bool acc_valid = false;
         uint32_t accfree_parity = 0;
         bool alive = true;
+        auto wait_all = [&](uint32_t bar, uint32_t parity) -> bool {
+            uint32_t ok = 1;
+            if (lane == 0) ok = bar_wait(bar, parity, abort_flag, p.status, false) ? 1u : 0u;
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            fence_after();
+            return ok != 0u;
+        };
         auto issue_E = [&](int64_t i) -> bool {
             const int s = (int)(i & 1);
             const uint32_t ph = (uint32_t)((i >> 1) & 1);
             TIC(tm_);
-            if (!bar_wait(BAR(B_YFULL0 + s), ph, abort_flag, p.status, false)) return false;
+            if (!wait_all(BAR(B_YFULL0 + s), ph)) return false;
             TOC(tm_, 12);
             TRACE(7, i);
-            fence_after();
-            const uint32_t yhi = smem_u32(smem + SM_Y + s * SM_YSTAGE), ylo = yhi + SM_YLO;
-            const uint32_t d = T_LOG + s * 64;
-            // The two small cross products go first: the accumulator truncates (toward zero) at every add, by up to one
-            // ulp of its CURRENT magnitude, so they are added while it is still small.
-            for (int ks = 0; ks < p.n_ks; ++ks)
-                mma_ss(d, make_desc(plo + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024),
-                       make_desc(yhi + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024), id_e, ks > 0);
-            for (int ks = 0; ks < p.n_ks; ++ks)
-                mma_ts(d, T_PHI + ks * 8, make_desc(ylo + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024), id_e, 1);
-            for (int ks = 0; ks < p.n_ks; ++ks)
-                mma_ts(d, T_PHI + ks * 8, make_desc(yhi + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024), id_e, 1);
-            mma_commit(BAR(B_LFULL0 + s));
+            if (elect_one()) {
+#ifdef FLASHGMM_DEBUG
+                if (p.dbg_y && rank == 0 && cluster_id == p.dbg_cluster && i == p.dbg_i) {
+                    const uint4* ys = reinterpret_cast<const uint4*>(smem + SM_Y + s * SM_YSTAGE);
+                    for (int q = 0; q < 4096; ++q) p.dbg_y[q] = ys[q];
+                }
+#endif
+                const uint32_t d = T_LOG + s * 64;
+                const uint64_t dyh = make_desc(y0 + s * SM_YSTAGE, 16, 1024);            // K-major views of the stage
+                const uint64_t dyl = make_desc(y0 + s * SM_YSTAGE + SM_YLO, 16, 1024);
+                // The two small cross products go first: the accumulator truncates (toward zero) at every add, by up to
+                // one ulp of its CURRENT magnitude, so they are added while it is still small.
+#pragma unroll
+                for (int ks = 0; ks < 16; ++ks)
+                    if (ks < n_ks) mma_ss(d, d_plo + (((ks >> 2) * 16384 + (ks & 3) * 32) >> 4),
+                                          dyh + (((ks >> 2) * 8192 + (ks & 3) * 32) >> 4), id_e, ks > 0);
+#pragma unroll
+                for (int ks = 0; ks < 16; ++ks)
+                    if (ks < n_ks) mma_ts(d, T_PHI + ks * 8, dyl + (((ks >> 2) * 8192 + (ks & 3) * 32) >> 4), id_e, 1);
+#pragma unroll
+                for (int ks = 0; ks < 16; ++ks)
+                    if (ks < n_ks) mma_ts(d, T_PHI + ks * 8, dyh + (((ks >> 2) * 8192 + (ks & 3) * 32) >> 4), id_e, 1);
+                mma_commit(BAR(B_LFULL0 + s));
+            }
+            __syncwarp();
             TOC(tm_, 13);
             TRACE(8, i);
             return true;
@@ -775,26 +811,41 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
             const int s = (int)(i & 1);
             const uint32_t ph = (uint32_t)((i >> 1) & 1);
             TIC(tm_);
-            if (!bar_wait(BAR(B_RREADY0 + s), ph, abort_flag, p.status, false)) return false;
+            if (!wait_all(BAR(B_RREADY0 + s), ph)) return false;
             TOC(tm_, 14);
             TRACE(9, i);
-            fence_after();
-            const uint32_t yhi = smem_u32(smem + SM_Y + s * SM_YSTAGE), ylo = yhi + SM_YLO;
-            // A operand layout in the logits buffer: points 0-31 -> columns [0,16) r_hi, [16,32) r_lo; points 32-63 -> +32
-            const uint32_t rbase = T_LOG + s * 64;
-            auto r_hi = [&](int ks) { return rbase + (ks >> 1) * 32 + (ks & 1) * 8; };
-            for (int ks = 0; ks < BN / 16; ++ks) {
-                mma_ts(T_ACC, r_hi(ks), make_desc(yhi + ks * 2048, 8192, 1024), id_m, acc_valid || ks > 0);
+            if (elect_one()) {
+                // A operand layout in the logits buffer: points 0-31 -> columns [0,16) r_hi, [16,32) r_lo; points 32-63 -> +32
+                const uint32_t rbase = T_LOG + s * 64;
+                const uint64_t dyh = make_desc(y0 + s * SM_YSTAGE, 8192, 1024);          // MN-major views of the stage
+                const uint64_t dyl = make_desc(y0 + s * SM_YSTAGE + SM_YLO, 8192, 1024);
+#pragma unroll
+                for (int ks = 0; ks < BN / 16; ++ks)
+                    mma_ts(T_ACC, rbase + (ks >> 1) * 32 + (ks & 1) * 8, dyh + ((ks * 2048) >> 4), id_m, (acc_valid || ks > 0) ? 1u : 0u);
+#pragma unroll
+                for (int ks = 0; ks < BN / 16; ++ks)
+                    mma_ts(T_ACC, rbase + (ks >> 1) * 32 + (ks & 1) * 8, dyl + ((ks * 2048) >> 4), id_m, 1);
+#pragma unroll
+                for (int ks = 0; ks < BN / 16; ++ks)
+                    mma_ts(T_ACC, rbase + (ks >> 1) * 32 + (ks & 1) * 8 + 16, dyh + ((ks * 2048) >> 4), id_m, 1);
+                mma_commit(BAR(B_YEMPTY0 + s));
             }
+            __syncwarp();
             acc_valid = true;
-            for (int ks = 0; ks < BN / 16; ++ks) mma_ts(T_ACC, r_hi(ks), make_desc(ylo + ks * 2048, 8192, 1024), id_m, 1);
-            for (int ks = 0; ks < BN / 16; ++ks) mma_ts(T_ACC, r_hi(ks) + 16, make_desc(yhi + ks * 2048, 8192, 1024), id_m, 1);
-            mma_commit(BAR(B_YEMPTY0 + s));
             TOC(tm_, 15);
             TRACE(10, i);
             return true;
         };
-        if (p.order == 0) {
+        // Hands the TMEM accumulators to the flushing softmax group and waits until they are free again.
+        auto flush_acc = [&]() -> bool {
+            if (elect_one()) mma_commit(BAR(B_ACCFULL));
+            __syncwarp();
+            if (!wait_all(BAR(B_ACCFREE), accfree_parity)) return false;
+            accfree_parity ^= 1;
+            acc_valid = false;
+            return true;
+        };
+        if ((p.order & 1) == 0) {
             // Issue order per pair of tiles: E(a) E(b) M(a) M(b).
             for (int64_t i = 0; i < ntl && alive; i += 2) {
                 const bool has2 = i + 1 < ntl;
@@ -804,13 +855,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                 if (alive && has2) alive = issue_M(i + 1);
                 if (!alive) break;
                 const int64_t pair_next = i + 2;
-                if ((pair_next % p.flush) == 0 || pair_next >= ntl) {
-                    mma_commit(BAR(B_ACCFULL));
-                    if (!bar_wait(BAR(B_ACCFREE), accfree_parity, abort_flag, p.status, false)) { alive = false; break; }
-                    accfree_parity ^= 1;
-                    fence_after();
-                    acc_valid = false;
-                }
+                if ((pair_next % p.flush) == 0 || pair_next >= ntl) alive = flush_acc();
             }
         } else {
             // Interleaved order E(0) E(1) | M(0) E(2) | M(1) E(3) | ...: M(i) must precede E(i+2) (two logits buffers, two
@@ -823,23 +868,34 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                 const bool pair_end = (i & 1) || (i + 1 == ntl);
                 const int64_t pair_next = (i | 1) + 1;
                 if (pair_end && ((pair_next % p.flush) == 0 || pair_next >= ntl)) {
-                    mma_commit(BAR(B_ACCFULL));
-                    if (!bar_wait(BAR(B_ACCFREE), accfree_parity, abort_flag, p.status, false)) { alive = false; break; }
-                    accfree_parity ^= 1;
-                    fence_after();
-                    acc_valid = false;
+                    alive = flush_acc();
+                    if (!alive) break;
                 }
                 if (i + 2 < ntl) alive = issue_E(i + 2);
             }
         }
-        // drain: every MMA issued by this thread has completed before TMEM is released
-        mma_commit(BAR(B_FINAL));
-        bar_wait(BAR(B_FINAL), 0, abort_flag, p.status, false);
+        // drain: every MMA issued by this warp has completed before TMEM is released
+        if (elect_one()) mma_commit(BAR(B_FINAL));
+        __syncwarp();
+        wait_all(BAR(B_FINAL), 0);
     }
 
     // teardown: everybody meets, peers are done with this CTA's shared memory, TMEM is released
     fence_before();
     __syncthreads();
+#ifdef FLASHGMM_DEBUG
+    if (p.dbg) {       // is the P_lo image in shared memory still what the prologue copied?
+        const uint4* src = reinterpret_cast<const uint4*>(p.plo_img + (size_t)rank * 65536);
+        const uint4* dst = reinterpret_cast<const uint4*>(smem + SM_PLO);
+        int bad = 0, first = -1;
+        for (int i = tid; i < 65536 / 16; i += NTHREADS) {
+            const uint4 a = __ldg(src + i), b = dst[i];
+            if (a.x != b.x || a.y != b.y || a.z != b.z || a.w != b.w) { ++bad; if (first < 0) first = i; }
+        }
+        if (bad && blockIdx.x < 8) printf("CTA %d thread %d: %d P_lo chunks differ, first chunk %d\n", (int)blockIdx.x, tid, bad, first);
+    }
+    __syncthreads();
+#endif
     if (warp == MMA_WARP) {
         fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512) : "memory");
@@ -1011,6 +1067,10 @@ long long* g_tc_clk = nullptr;
 long long* g_tc_trace = nullptr;
 extern "C" void gmm_debug_set_trace(long long* p) { g_tc_trace = p; }
 extern "C" void gmm_debug_set_buffer(float* p) { g_tc_debug = p; }
+int g_tc_dbg_cluster = 0, g_tc_dbg_i = 0;
+uint4* g_tc_dbg_y = nullptr;
+extern "C" void gmm_debug_set_ybuf(void* p) { g_tc_dbg_y = static_cast<uint4*>(p); }
+extern "C" void gmm_debug_set_select(int cluster, int i) { g_tc_dbg_cluster = cluster; g_tc_dbg_i = i; }
 extern "C" void gmm_debug_set_clk(long long* p) { g_tc_clk = p; }
 #endif
 
@@ -1068,6 +1128,7 @@ cudaError_t launch_em_tc(cudaStream_t s, const float* X, int64_t n, int D, int K
     p.xg = static_cast<XSlot*>(tb.xg); p.xl = static_cast<XSlot*>(tb.xl);
 #ifdef FLASHGMM_DEBUG
     p.dbg = g_tc_debug;
+    p.dbg_cluster = g_tc_dbg_cluster; p.dbg_i = g_tc_dbg_i; p.dbg_y = g_tc_dbg_y;
     p.dbg_clk = g_tc_clk;
     p.dbg_trace = g_tc_trace;
 #endif

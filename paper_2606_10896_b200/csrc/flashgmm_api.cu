@@ -344,7 +344,10 @@ int gmm_create(gmm_ctx** out, int device, void* cuda_stream) {
     ctx->stream = static_cast<cudaStream_t>(cuda_stream);
     if (const char* e = std::getenv("GMM_TC_COND_LIMIT")) ctx->tc_cond_limit = (float)std::atof(e);
     if (const char* e = std::getenv("GMM_TC_FLUSH")) ctx->tc_flush = std::atoi(e);
-    if (const char* e = std::getenv("GMM_TC_ORDER")) tc_set_order(std::atoi(e));
+    {   // the issue order is process-wide: every create sets it, so a context never inherits an earlier context's choice
+        const char* e = std::getenv("GMM_TC_ORDER");
+        tc_set_order(e ? std::atoi(e) : 1);
+    }
     *out = ctx;
     return GMM_OK;
 }

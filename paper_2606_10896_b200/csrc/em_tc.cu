@@ -794,12 +794,15 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                 for (int ks = 0; ks < 16; ++ks)
                     if (ks < n_ks) mma_ss(d, d_plo + (((ks >> 2) * 16384 + (ks & 3) * 32) >> 4),
                                           dyh + (((ks >> 2) * 8192 + (ks & 3) * 32) >> 4), id_e, ks > 0);
+                TRACE(11, i);
 #pragma unroll
                 for (int ks = 0; ks < 16; ++ks)
                     if (ks < n_ks) mma_ts(d, T_PHI + ks * 8, dyl + (((ks >> 2) * 8192 + (ks & 3) * 32) >> 4), id_e, 1);
+                TRACE(12, i);
 #pragma unroll
                 for (int ks = 0; ks < 16; ++ks)
                     if (ks < n_ks) mma_ts(d, T_PHI + ks * 8, dyh + (((ks >> 2) * 8192 + (ks & 3) * 32) >> 4), id_e, 1);
+                TRACE(13, i);
                 mma_commit(BAR(B_LFULL0 + s));
             }
             __syncwarp();

@@ -10,6 +10,7 @@
 // log2 z = c2 - sum_d w2 (x - mu)^2, so the exponential is a bare ex2.
 #include "internal.cuh"
 #include <math_constants.h>
+#include <stdint.h>
 
 namespace fg {
 
@@ -48,26 +49,54 @@ __device__ __forceinline__ void tile_quadratic(TileSmem& sm, const float* __rest
     for (int a = 0; a < 4; ++a)
 #pragma unroll
         for (int b = 0; b < 4; ++b) q[a][b] = (ACC)0;
+    // Staging: the tile's next 32 dimensions are fetched into registers (16-byte loads: eight consecutive threads read
+    // 128 bytes of one row) while the current 32 are being computed from shared memory, so the load latency is hidden
+    // behind the arithmetic instead of being exposed at every stage.
+    const bool vec = (D % 4 == 0) && (((reinterpret_cast<uintptr_t>(X) | reinterpret_cast<uintptr_t>(mu) |
+                                        reinterpret_cast<uintptr_t>(w2)) & 15) == 0);
+    float4 px[2], pm[2], pw[2];
+    auto fetch = [&](int d0) {
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const int e4 = tid + j * NTHREADS, r = e4 >> 3, d = d0 + (e4 & 7) * 4;
+            const int64_t row = row0 + r;
+            const int k = k0 + r;
+            px[j] = pm[j] = pw[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (vec && d + 4 <= D) {
+                if (row < n) px[j] = __ldg(reinterpret_cast<const float4*>(X + row * D + d));
+                if (k < K) {
+                    pm[j] = __ldg(reinterpret_cast<const float4*>(mu + (size_t)k * D + d));
+                    pw[j] = __ldg(reinterpret_cast<const float4*>(w2 + (size_t)k * D + d));
+                }
+            } else {
+                float xv[4] = {0.f, 0.f, 0.f, 0.f}, mv[4] = {0.f, 0.f, 0.f, 0.f}, wv[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int t = 0; t < 4; ++t)
+                    if (d + t < D) {
+                        if (row < n) xv[t] = __ldg(X + row * D + d + t);
+                        if (k < K) {
+                            mv[t] = __ldg(mu + (size_t)k * D + d + t);
+                            wv[t] = __ldg(w2 + (size_t)k * D + d + t);
+                        }
+                    }
+                px[j] = make_float4(xv[0], xv[1], xv[2], xv[3]);
+                pm[j] = make_float4(mv[0], mv[1], mv[2], mv[3]);
+                pw[j] = make_float4(wv[0], wv[1], wv[2], wv[3]);
+            }
+        }
+    };
+    fetch(0);
     for (int d0 = 0; d0 < D; d0 += DCH) {
         __syncthreads();
 #pragma unroll
-        for (int j = 0; j < (TP * DCH) / NTHREADS; ++j) {
-            const int e = tid + j * NTHREADS, r = e >> 5, c = e & 31, d = d0 + c;
-            const int64_t row = row0 + r;
-            const int k = k0 + r;
-            float xv = 0.f, mv = 0.f, wv = 0.f;
-            if (d < D) {
-                if (row < n) xv = __ldg(X + row * D + d);
-                if (k < K) {
-                    mv = __ldg(mu + (size_t)k * D + d);
-                    wv = __ldg(w2 + (size_t)k * D + d);
-                }
-            }
-            sm.xs[c][r] = xv;
-            sm.ms[c][r] = mv;
-            sm.ws[c][r] = wv;
+        for (int j = 0; j < 2; ++j) {
+            const int e4 = tid + j * NTHREADS, r = e4 >> 3, c = (e4 & 7) * 4;
+            sm.xs[c][r] = px[j].x; sm.xs[c + 1][r] = px[j].y; sm.xs[c + 2][r] = px[j].z; sm.xs[c + 3][r] = px[j].w;
+            sm.ms[c][r] = pm[j].x; sm.ms[c + 1][r] = pm[j].y; sm.ms[c + 2][r] = pm[j].z; sm.ms[c + 3][r] = pm[j].w;
+            sm.ws[c][r] = pw[j].x; sm.ws[c + 1][r] = pw[j].y; sm.ws[c + 2][r] = pw[j].z; sm.ws[c + 3][r] = pw[j].w;
         }
         __syncthreads();
+        if (d0 + DCH < D) fetch(d0 + DCH);
         float part[4][4];
 #pragma unroll
         for (int a = 0; a < 4; ++a)
@@ -250,7 +279,7 @@ constexpr int LDX = FP32_MSTEP_DC + 4;      // X tile row stride
 constexpr size_t MSTEP_SMEM = sizeof(TileSmem) + (size_t)TP * LDR * 4 + (size_t)TP * LDX * 4;
 
 template <typename ACC>
-__global__ void __launch_bounds__(NTHREADS)
+__global__ void __launch_bounds__(NTHREADS, sizeof(ACC) == 4 ? 2 : 1)      // float logits: two CTAs per SM
 mstep_kernel(const float* __restrict__ X, int64_t n, int D, int K, const float* __restrict__ mu,
              const float* __restrict__ w2, const double* __restrict__ c2, const double* __restrict__ logZ2,
              float* __restrict__ partials) {
@@ -510,9 +539,27 @@ Fp32Plan fp32_plan(int D, int K) {
     p.d_chunks = (D + FP32_MSTEP_DC - 1) / FP32_MSTEP_DC;
     p.wide = D > FP32_MSTEP_DC;
     // wide shapes: one CTA loops over the D slices itself (one resident CTA per SM: float64 logits are register-hungry)
-    const int per = p.wide ? p.comp_blocks : p.comp_blocks * p.d_chunks;
-    const int target = p.wide ? 148 : FP32_TARGET_CTAS;
-    p.splits = (target + per - 1) / per;
+    if (p.wide) {
+        // One resident CTA per SM: pick the number of point splits whose grid fills whole waves of 148 SMs best (a
+        // grid of 1.3 waves leaves most SMs idle through the second one), among those whose float64 partials stay
+        // within 256 MB.
+        const size_t per_split = ((size_t)K + 2 * (size_t)K * D) * sizeof(double);
+        int max_sp = (int)(((size_t)256 << 20) / per_split);
+        if (max_sp < 1) max_sp = 1;
+        if (max_sp > 148) max_sp = 148;
+        int best = 1;
+        double best_eff = 0.0;
+        for (int sp = 1; sp <= max_sp; ++sp) {
+            const int ctas = p.comp_blocks * sp;
+            const int waves = (ctas + 147) / 148;
+            const double eff = (double)ctas / (148.0 * waves);
+            if (eff > best_eff + 1e-9) { best_eff = eff; best = sp; }
+        }
+        p.splits = best;
+        return p;
+    }
+    const int per = p.comp_blocks * p.d_chunks;
+    p.splits = (FP32_TARGET_CTAS + per - 1) / per;
     if (p.splits < 1) p.splits = 1;
     return p;
 }

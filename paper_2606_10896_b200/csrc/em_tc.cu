@@ -195,7 +195,9 @@ __device__ __forceinline__ bool xslot_wait(const XSlot* q, uint32_t tag, float& 
 }
 
 // Bounded poll of the CL slots of one point (stride 64 slots between source CTAs): all outstanding loads are issued
-// together, so one round costs one L2 round trip.
+// together, so one round costs one L2 round trip.  Called by a whole warp, one point per lane; the warp leaves the loop
+// TOGETHER (when every lane has all its slots): lanes that left at different rounds would run the code that follows
+// once per group of lanes, which cost more than the wait itself.
 __device__ __forceinline__ bool xslot_wait_all(const XSlot* q, int CL, uint32_t tag, float2 (&e)[8], volatile int* abort_flag,
                                                int* status) {
     uint32_t pending = (CL >= 32) ? 0xffffffffu : ((1u << CL) - 1u);
@@ -213,17 +215,18 @@ __device__ __forceinline__ bool xslot_wait_all(const XSlot* q, int CL, uint32_t 
                 e[c] = make_float2(__uint_as_float(v[c][0]), __uint_as_float(v[c][2]));
                 pending &= ~(1u << c);
             }
-        if (pending == 0u) return true;
-        if (*abort_flag) return false;
+        if (__all_sync(0xffffffffu, pending == 0u)) return true;
+        bool give_up = *abort_flag != 0;
         if ((it & 15) == 15) {
             const unsigned long long now = gtime();
             if (t0 == 0) t0 = now;
             else if (now - t0 > WAIT_LIMIT_NS) {
                 *abort_flag = 1;
                 atomicOr(status, ST_TIMEOUT);
-                return false;
+                give_up = true;
             }
         }
+        if (__any_sync(0xffffffffu, give_up)) return false;
     }
 }
 
@@ -420,7 +423,11 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
         XSlot* xg = p.xg + (size_t)cluster_id * 4 * p.CL * 64;             // [4][CL][64] ring of exchange slots
         XSlot* xl = p.xl + (size_t)cluster_id * 4 * p.CL * 256;            // [4][CL][4 warps][64]: lower bounds (ill-conditioned mode)
         float nk_acc = 0.f;
-        double ll_acc = 0.0;
+        // log2 Z of this lane's points (rank 0, first warp of the group): a compensated fp32 sum, formed AFTER the tile's
+        // responsibilities were handed over, so that neither float64 arithmetic nor the logarithm sits on the path that
+        // the whole group of CTAs waits on
+        float ll_s = 0.f, ll_c = 0.f, ll_m = 0.f, ll_z = 1.f;
+        bool ll_have = false;
         // partial layout [group][column][component]: the 32 lanes of a warp touch 32 consecutive doubles; every address
         // belongs to exactly one thread of the grid, so the reductions below are deterministic
         const size_t pstride = (size_t)p.CL * 128;
@@ -582,12 +589,15 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
 #pragma unroll
                 for (int c = 0; c < 8; ++c)
                     Z += (e[c].x == -CUDART_INF_F) ? 0.f : e[c].y * fast_ex2(e[c].x - mi_safe);
+                TOC(tk_, 19);
                 const bool valid = pt < nvalid;
-                const float inv = (valid && Z > 0.f) ? (RSCALE / Z) : 0.f;
+                const float inv = (valid && Z > 0.f) ? __fdividef(RSCALE, Z) : 0.f;
 #pragma unroll
                 for (int w = 0; w < 4; ++w)
                     fac[w * 32 + pt] = (w4[w].x == -CUDART_INF_F) ? 0.f : fast_ex2(w4[w].x - mi_safe) * inv;
-                if (rank == 0 && valid) ll_acc += (double)(mi + log2f(Z));
+                TOC(tk_, 20);
+                ll_have = rank == 0 && valid;
+                ll_m = mi; ll_z = Z;
             }
             if (gtid == 0) decision_s[grp] = *abort_flag;
             TOC(tk_, 5);
@@ -624,6 +634,13 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
             bar_arrive(BAR(B_RREADY0 + s));
             TOC(tk_, 7);
             if (gtid == 0) TRACE(4, i);
+            if (gtid < 32 && ll_have) {              // two-sum: (ll_s, ll_c) += log2 Z_i exactly to fp32 pair precision
+                const float v = ll_m + log2f(ll_z);
+                const float t = ll_s + v;
+                const float bp = t - ll_s;
+                ll_c += (ll_s - (t - bp)) + (v - bp);
+                ll_s = t;
+            }
 
             // periodic flush of the TMEM accumulators into float64 partials, by group 1, after the second tile of a pair
             // (or the last tile); the flush index (hence the barrier parity) follows from the tile index alone
@@ -653,7 +670,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
         }
         if (rank == 0) {
             double* lls = reinterpret_cast<double*>(smem + SM_LL) + grp * 32;
-            if (gtid < 32) lls[gtid] = ll_acc;
+            if (gtid < 32) lls[gtid] = (double)ll_s + (double)ll_c;
             named_bar_sync(5 + grp, 128);
             if (gtid == 0) {
                 double sum = 0.0;

@@ -136,6 +136,13 @@ __device__ __forceinline__ void bar_init(uint32_t bar, uint32_t count) {
 __device__ __forceinline__ void bar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+// Non-blocking test of an mbarrier phase.
+__device__ __forceinline__ bool bar_test(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0u;
+}
 // ---- exchange between the CTAs of a group through global memory (L2).  A slot is two 64-bit words {value, tag}: each
 //      word is written and read as one unit, so a reader that sees the expected tag in both words has both values.
 //      Slots form a ring of 4 per (group, source CTA): a CTA writes tile i+4 only after it has finished tile i+2, which
@@ -448,6 +455,22 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
             TOC(tk_, 0);
             if (gtid == 0) TRACE(0, i);
             fence_after();
+#ifdef FLASHGMM_DEBUG
+            if (p.order & 4) {                // what-if timing only: no softmax work at all
+                fence_before();
+                bar_arrive(BAR(B_RREADY0 + s));
+                const bool pe = (i & 1) || (i + 1 == ntl);
+                const int64_t pn = (i | 1) + 1;
+                if (grp == 1 && pe && ((pn % p.flush) == 0 || pn >= ntl)) {
+                    const uint32_t fpar = (uint32_t)(((pn - 1) / p.flush) & 1);
+                    bar_wait(BAR(B_ACCFULL), fpar, abort_flag, p.status, false);
+                    fence_after();
+                    fence_before();
+                    bar_arrive(BAR(B_ACCFREE));
+                }
+                continue;
+            }
+#endif
             float l[32];
             {
                 uint32_t v0[32];
@@ -578,6 +601,12 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                 xslot_write(ring + rank * 64, mc, sc, tag);
                 TOC(tk_, 3);
                 float2 e[8];
+#ifdef FLASHGMM_DEBUG
+                if (p.order & 64) {           // what-if timing only (results are wrong): do not wait for the peers
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) e[c] = make_float2(mc, sc);
+                } else
+#endif
                 if (!xslot_wait_all(ring, p.CL, tag, e, abort_flag, p.status)) alive = false;
                 float mi = -CUDART_INF_F;
 #pragma unroll
@@ -746,6 +775,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
             }
             TOC(tt_, 10);
             if (tau == 0) TRACE(5, i);
+#ifdef FLASHGMM_DEBUG
+            if (!(p.order & 8))               // what-if timing only: no shared-memory stores
+#endif
 #pragma unroll
             for (int n = 0; n < NU; ++n) {
                 const int u = tau + n * TR_THREADS;
@@ -788,11 +820,11 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
             fence_after();
             return ok != 0u;
         };
-        auto issue_E = [&](int64_t i) -> bool {
+        auto issue_E = [&](int64_t i, bool seen = false) -> bool {
             const int s = (int)(i & 1);
             const uint32_t ph = (uint32_t)((i >> 1) & 1);
             TIC(tm_);
-            if (!wait_all(BAR(B_YFULL0 + s), ph)) return false;
+            if (!seen && !wait_all(BAR(B_YFULL0 + s), ph)) return false;
             TOC(tm_, 12);
             TRACE(7, i);
             if (elect_one()) {
@@ -803,6 +835,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                 }
 #endif
                 const uint32_t d = T_LOG + s * 64;
+#ifdef FLASHGMM_DEBUG
+                if (!(p.order & 16)) {        // what-if timing only: no E-step MMAs
+#endif
                 const uint64_t dyh = make_desc(y0 + s * SM_YSTAGE, 16, 1024);            // K-major views of the stage
                 const uint64_t dyl = make_desc(y0 + s * SM_YSTAGE + SM_YLO, 16, 1024);
                 // The two small cross products go first: the accumulator truncates (toward zero) at every add, by up to
@@ -820,6 +855,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                 for (int ks = 0; ks < 16; ++ks)
                     if (ks < n_ks) mma_ts(d, T_PHI + ks * 8, dyh + (((ks >> 2) * 8192 + (ks & 3) * 32) >> 4), id_e, 1);
                 TRACE(13, i);
+#ifdef FLASHGMM_DEBUG
+                }
+#endif
                 mma_commit(BAR(B_LFULL0 + s));
             }
             __syncwarp();
@@ -827,16 +865,19 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
             TRACE(8, i);
             return true;
         };
-        auto issue_M = [&](int64_t i) -> bool {
+        auto issue_M = [&](int64_t i, bool seen = false) -> bool {
             const int s = (int)(i & 1);
             const uint32_t ph = (uint32_t)((i >> 1) & 1);
             TIC(tm_);
-            if (!wait_all(BAR(B_RREADY0 + s), ph)) return false;
+            if (!seen && !wait_all(BAR(B_RREADY0 + s), ph)) return false;
             TOC(tm_, 14);
             TRACE(9, i);
             if (elect_one()) {
                 // A operand layout in the logits buffer: points 0-31 -> columns [0,16) r_hi, [16,32) r_lo; points 32-63 -> +32
                 const uint32_t rbase = T_LOG + s * 64;
+#ifdef FLASHGMM_DEBUG
+                if (!(p.order & 32)) {        // what-if timing only: no M-step MMAs
+#endif
                 const uint64_t dyh = make_desc(y0 + s * SM_YSTAGE, 8192, 1024);          // MN-major views of the stage
                 const uint64_t dyl = make_desc(y0 + s * SM_YSTAGE + SM_YLO, 8192, 1024);
 #pragma unroll
@@ -848,6 +889,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
 #pragma unroll
                 for (int ks = 0; ks < BN / 16; ++ks)
                     mma_ts(T_ACC, rbase + (ks >> 1) * 32 + (ks & 1) * 8 + 16, dyh + ((ks * 2048) >> 4), id_m, 1);
+#ifdef FLASHGMM_DEBUG
+                }
+#endif
                 mma_commit(BAR(B_YEMPTY0 + s));
             }
             __syncwarp();
@@ -865,7 +909,48 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
             acc_valid = false;
             return true;
         };
-        if ((p.order & 1) == 0) {
+        if ((p.order & 3) == 2) {
+            // Dynamic order: E(j) needs its Y stage (and M(j-2) issued, which frees that stage and logits buffer), M(i)
+            // needs the responsibilities of tile i; the two are independent, so whichever is ready first is issued.
+            // With a fixed order the warp sat in the wait for the refill of E(i+2)'s stage while M(i+1) was ready.
+            int64_t next_e = 0, next_m = 0;
+            unsigned long long t0 = 0;
+            int spins = 0;
+            while (next_m < ntl && alive) {
+                uint32_t act = 0;                                   // 1: E(next_e)   2: M(next_m)   3: give up
+                if (lane == 0) {
+                    if (next_e < ntl && next_e < next_m + 2 &&
+                        bar_test(BAR(B_YFULL0 + (int)(next_e & 1)), (uint32_t)((next_e >> 1) & 1))) act = 1;
+                    else if (next_m < next_e && bar_test(BAR(B_RREADY0 + (int)(next_m & 1)), (uint32_t)((next_m >> 1) & 1))) act = 2;
+                    else if (*abort_flag) act = 3;
+                    else if ((++spins & 63) == 0) {
+                        const unsigned long long now = gtime();
+                        if (t0 == 0) t0 = now;
+                        else if (now - t0 > WAIT_LIMIT_NS) {
+                            *abort_flag = 1;
+                            atomicOr(p.status, ST_TIMEOUT);
+                            act = 3;
+                        }
+                    }
+                }
+                act = __shfl_sync(0xffffffffu, act, 0);
+                if (act == 0) continue;
+                if (act == 3) { alive = false; break; }
+                t0 = 0; spins = 0;
+                fence_after();
+                if (act == 1) {
+                    alive = issue_E(next_e, true);
+                    ++next_e;
+                } else {
+                    const int64_t i = next_m;
+                    alive = issue_M(i, true);
+                    ++next_m;
+                    const bool pair_end = (i & 1) || (i + 1 == ntl);
+                    const int64_t pair_next = (i | 1) + 1;
+                    if (alive && pair_end && ((pair_next % p.flush) == 0 || pair_next >= ntl)) alive = flush_acc();
+                }
+            }
+        } else if ((p.order & 1) == 0) {
             // Issue order per pair of tiles: E(a) E(b) M(a) M(b).
             for (int64_t i = 0; i < ntl && alive; i += 2) {
                 const bool has2 = i + 1 < ntl;

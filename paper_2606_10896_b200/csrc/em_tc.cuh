@@ -34,7 +34,7 @@ struct TcBuffers {
 };
 
 bool tc_supports(int D, int K);
-void tc_set_order(int o);   // MMA issue order: 0 = pairs E E M M, 1 = interleaved M(i) E(i+2)
+void tc_set_order(int o);   // MMA issue order: 0 = pairs E E M M, 1 = interleaved M(i) E(i+2) (default), 2 = whichever of E(i+2), M(i+1) is ready first
 TcPlan tc_plan(int D, int K, int num_sms);
 size_t tc_scratch_bytes(int D, int K);
 cudaError_t tc_max_clusters(int D, int K, int* out);

@@ -104,11 +104,12 @@ def test_config2_cut_teacher_forced(fg, ctx):
     _teacher_forced(fg, ctx, synth.sample_host(spec), spec, 3)
 
 
-@pytest.mark.parametrize("order", ["0", "1"])
+@pytest.mark.parametrize("order", ["0", "1", "2"])
 def test_tensor_ill_conditioned_mode_under_both_issue_orders(fg, order, monkeypatch):
     # From the second iteration on, N=3000 < 3K leaves most components collapsed onto single points at the variance
     # floor: the tensor path runs its exact-recomputation protocol.  Three point tiles per group of CTAs, so the
-    # interleaved order issues E(2) between M(0) and M(1).  Both MMA issue orders must give the same, correct statistics.
+    # interleaved order issues E(2) between M(0) and M(1).  Every MMA issue order (pairs, interleaved, dynamic) must give
+    # the same, correct statistics.
     monkeypatch.setenv("GMM_TC_ORDER", order)
     spec = synth.CONFIGS[2].with_n(3000)
     with fg.Context(0) as c:

@@ -501,18 +501,30 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                 // valid lower bound (and for a warp without flagged lanes it is the maximum itself)
                 const uint32_t tag = (uint32_t)(i + 1);
                 XSlot* ring = xl + (size_t)(i & 3) * p.CL * 256 + p0;
-                xslot_write(ring + (rank * 4 + wq) * 64 + lane, red - emax_w, 0.f, tag);     // publish: no barrier, no wait
+                const float lb_own = red - emax_w;                      // this warp's lower bound for point `lane`
+                uint32_t mlo = 0;
                 if (emax_w > 0.f) {
-                    gather[lane] = red - emax_w;
-                    __syncwarp();
-                    const int kglob = (int)rank * 128 + kloc;
-                    uint32_t mlo = 0;
-                    if (illb > 0.f) {
+#ifdef FLASHGMM_DEBUG
+                    if (p.dbg_clk && blockIdx.x == 0 && lane == 0) atomicAdd((unsigned long long*)&p.dbg_clk[26], 1ull);
+                    if (p.dbg_clk && blockIdx.x == 0 && i == 0 && illb > 0.f) atomicAdd((unsigned long long*)&p.dbg_clk[27], 1ull);
+#endif
+                    // Local filter, by shuffles (no shared memory, no warp barrier: a barrier here would also wait for
+                    // global stores in flight): bit j of mlo = point j of this lane's component may matter.
+                    const float reach = (illb > 0.f) ? illb + ILL_MARGIN : -CUDART_INF_F;
 #pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (j < nvalid && l[j] + illb >= gather[j] - ILL_MARGIN) mlo |= 1u << j;
+                    for (int j = 0; j < 32; ++j) {
+                        const float lbj = __shfl_sync(0xffffffffu, lb_own, j);
+                        if (j < nvalid && l[j] + reach >= lbj) mlo |= 1u << j;
                     }
+                }
+                // publish AFTER the filter: peers read these slots only for the rare pairs that survive their own filter,
+                // and a global store in flight makes the next warp-level barrier wait for it
+                xslot_write(ring + (rank * 4 + wq) * 64 + lane, lb_own, 0.f, tag);
+                TOC(tk_, 28);
+                if (emax_w > 0.f) {
+                    const int kglob = (int)rank * 128 + kloc;
                     bool fixed_any = false;
+                    TOC(tk_, 29);
                     for (;;) {
                         const uint32_t ballot = __ballot_sync(0xffffffffu, mlo != 0u);
                         if (ballot == 0u) break;
@@ -534,7 +546,13 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                         }
 #pragma unroll
                         for (int o = 16; o > 0; o >>= 1) lbv = fmaxf(lbv, __shfl_xor_sync(0xffffffffu, lbv, o));
+#ifdef FLASHGMM_DEBUG
+                        if (p.dbg_clk && blockIdx.x == 0 && lane == 0) atomicAdd((unsigned long long*)&p.dbg_clk[24], 1ull);
+#endif
                         if (ub >= lbv - ILL_MARGIN) {
+#ifdef FLASHGMM_DEBUG
+                            if (p.dbg_clk && blockIdx.x == 0 && lane == 0) atomicAdd((unsigned long long*)&p.dbg_clk[25], 1ull);
+#endif
                             const float* xr = p.X + (row0 + p0 + j) * p.D;
                             const float* mr = p.mu + (size_t)kk * p.D;
                             const float* wr = p.w2 + (size_t)kk * p.D;
@@ -556,6 +574,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                         if (lane == src) mlo &= ~(1u << j);
                     }
                     __syncwarp();
+                    TOC(tk_, 30);
                     if (fixed_any) warp_reduce_scatter32<true>(l, red, lane);      // maxima with the corrected logits
                 }
             }

@@ -20,8 +20,11 @@
 // MN-major by the M-step), exchange buffers, barriers.
 //
 // Warp roles: warps 0-7 softmax (two warpgroups, each taking 32 of a tile's 64 points; warp w owns TMEM lanes
-// 32 (w mod 4) ...), warps 8-14 load X with coalesced 16-byte loads and build the Y planes, warp 15 issues the MMAs.  Every wait is bounded by a wall-clock limit; on expiry the CTA sets
-// ST_TIMEOUT, all roles leave their loops, TMEM is freed and the kernel returns.
+// 32 (w mod 4) ...), warps 8-14 load X with coalesced 16-byte loads and build the Y planes, warp 15 issues the MMAs: the
+// whole warp runs the issue loop convergently, lane 0 does the waits and broadcasts their outcome, one elected lane
+// issues (descriptors = hoisted base + immediate offset, loops unrolled) and commits.  Three issue orders exist (pairs,
+// interleaved = default, whichever-is-ready); all give identical results.  Every wait is bounded by a wall-clock limit;
+// on expiry the CTA sets ST_TIMEOUT, all roles leave their loops, TMEM is freed and the kernel returns.
 #include "internal.cuh"
 #include "em_tc.cuh"
 

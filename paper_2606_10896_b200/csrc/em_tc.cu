@@ -669,6 +669,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                     const float2 b01 = __half22float2(h01), b23 = __half22float2(h23);
                     const __half2 g01 = __floats2half2_rn(r0 - b01.x, r1 - b01.y), g23 = __floats2half2_rn(r2 - b23.x, r3 - b23.y);
                     const float2 c01 = __half22float2(g01), c23 = __half22float2(g23);
+                    // N_k must be the sum of exactly the weights the M-step uses (hi + lo): responsibilities too small for
+                    // fp16 vanish from S1 and S2, and a dying component whose N_k still counted them would get mu = S1 / N_k
+                    // pulled toward zero instead of staying a weighted mean
                     nsum += ((b01.x + c01.x) + (b01.y + c01.y)) + ((b23.x + c23.x) + (b23.y + c23.y));
                     hi[j / 2] = *reinterpret_cast<const uint32_t*>(&h01);
                     hi[j / 2 + 1] = *reinterpret_cast<const uint32_t*>(&h23);
@@ -736,6 +739,10 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
         // into its four fp16 planes in registers BEFORE the wait for the stage, so that only the shared-memory stores
         // sit between the release of a stage and its next use.
         const int tau = tid - 256;
+        // a thread's eight dimensions never change (224 is a multiple of 16): their scales and shifts stay in registers
+        float sdr[8], kpr[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { sdr[j] = sd_s[(tau & 15) * 8 + j]; kpr[j] = kap_s[(tau & 15) * 8 + j]; }
         const bool vec_ok = (p.D % 4 == 0) && ((reinterpret_cast<uintptr_t>(p.X) & 15) == 0);
         constexpr int NU = 5;                               // ceil(1024 / 224)
         for (int64_t i = 0; i < ntl; ++i) {
@@ -766,15 +773,14 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
             uint4 vxh[NU], vxl[NU], vqh[NU], vql[NU];
 #pragma unroll
             for (int n = 0; n < NU; ++n) {
-                const int d0 = ((tau + n * TR_THREADS) & 15) * 8;
                 const float x[8] = {xa[n].x, xa[n].y, xa[n].z, xa[n].w, xb[n].x, xb[n].y, xb[n].z, xb[n].w};
                 uint32_t xh[4], xl[4], qh[4], ql[4];
 #pragma unroll
                 for (int j = 0; j < 8; j += 2) {
-                    float u0 = x[j] * sd_s[d0 + j], u1 = x[j + 1] * sd_s[d0 + j + 1];
+                    float u0 = x[j] * sdr[j], u1 = x[j + 1] * sdr[j + 1];
                     u0 = fminf(fmaxf(u0, -240.f), 240.f);
                     u1 = fminf(fmaxf(u1, -240.f), 240.f);
-                    const float q0 = fmaf(u0, u0, kap_s[d0 + j]), q1 = fmaf(u1, u1, kap_s[d0 + j + 1]);
+                    const float q0 = fmaf(u0, u0, kpr[j]), q1 = fmaf(u1, u1, kpr[j + 1]);
                     const __half2 h = __floats2half2_rn(u0, u1);
                     const float2 hf = __half22float2(h);
                     const __half2 g2 = __floats2half2_rn(u0 - hf.x, u1 - hf.y);

@@ -381,10 +381,10 @@ mstep_kernel(const float* __restrict__ X, int64_t n, int D, int K, const float* 
 // of D, accumulating each slice over the whole batch in registers and adding it to this CTA's own rows of a float64
 // partial in global memory (no other CTA touches them: deterministic, no atomics).  The E-step is thus recomputed once
 // per point and component, not once per slice of D.
-constexpr int WT = 6;
+constexpr int WT = 3;
 constexpr size_t MSTEP_WIDE_SMEM = sizeof(TileSmem) + (size_t)WT * TP * LDR * 4 + (size_t)TP * LDX * 4;
 
-__global__ void __launch_bounds__(NTHREADS)
+__global__ void __launch_bounds__(NTHREADS, 2)
 mstep_wide_kernel(const float* __restrict__ X, int64_t n, int D, int K, const float* __restrict__ mu,
                   const float* __restrict__ w2, const double* __restrict__ c2, const double* __restrict__ logZ2,
                   double* __restrict__ partials) {
@@ -540,19 +540,19 @@ Fp32Plan fp32_plan(int D, int K) {
     p.wide = D > FP32_MSTEP_DC;
     // wide shapes: one CTA loops over the D slices itself (one resident CTA per SM: float64 logits are register-hungry)
     if (p.wide) {
-        // One resident CTA per SM: pick the number of point splits whose grid fills whole waves of 148 SMs best (a
+        // Two resident CTAs per SM: pick the number of point splits whose grid fills whole waves of 296 CTAs best (a
         // grid of 1.3 waves leaves most SMs idle through the second one), among those whose float64 partials stay
         // within 256 MB.
         const size_t per_split = ((size_t)K + 2 * (size_t)K * D) * sizeof(double);
         int max_sp = (int)(((size_t)256 << 20) / per_split);
         if (max_sp < 1) max_sp = 1;
-        if (max_sp > 148) max_sp = 148;
+        if (max_sp > 296) max_sp = 296;
         int best = 1;
         double best_eff = 0.0;
         for (int sp = 1; sp <= max_sp; ++sp) {
             const int ctas = p.comp_blocks * sp;
-            const int waves = (ctas + 147) / 148;
-            const double eff = (double)ctas / (148.0 * waves);
+            const int waves = (ctas + 295) / 296;
+            const double eff = (double)ctas / (296.0 * waves);
             if (eff > best_eff + 1e-9) { best_eff = eff; best = sp; }
         }
         p.splits = best;

@@ -155,7 +155,9 @@ int gmm_em_step_static(int device, void* cuda_stream, const float* X, int64_t N,
                        const float* pi, const float* mu, const float* var,
                        double* Nk, double* S1, double* S2, double* loglik);
 
-/* Bytes of device scratch a context holds for shape (D, K); independent of N. */
+/* Bytes of device scratch a context in GMM_PATH_AUTO holds for shape (D, K); independent of N.  Where the tensor
+ * path runs (see gmm_auto_path) this includes 512 MiB for the fp16 planes of one launch-sized piece of the data;
+ * forcing GMM_PATH_TENSOR on a shape AUTO sends to the FP32 path adds the same 512 MiB. */
 size_t gmm_scratch_bytes(int D, int K);
 
 /* Instrumentation.  Kernel launches enqueued by this context since creation (or the last reset). */

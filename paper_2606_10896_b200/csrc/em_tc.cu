@@ -28,6 +28,7 @@
 #include "internal.cuh"
 #include "em_tc.cuh"
 
+#include <cuda.h>
 #include <cuda_fp16.h>
 #ifdef FLASHGMM_DEBUG
 #include <cstdio>
@@ -41,7 +42,7 @@ namespace {
 constexpr int BN = TC_BN;                 // points per tile
 constexpr int NTHREADS = 512;          // 8 softmax warps, 7 transform warps, 1 MMA warp (16 warps: 128 registers each)
 constexpr int MMA_WARP = 15;
-constexpr int TR_THREADS = 224;
+constexpr int PRODUCER_WARP = 8;
 constexpr float RSCALE = TC_RSCALE;
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 constexpr float ILL_MARGIN = 40.f;     // log2 units: a logit more than this below the best one is negligible (2^-40)
@@ -138,6 +139,20 @@ __device__ __forceinline__ void bar_init(uint32_t bar, uint32_t count) {
 }
 __device__ __forceinline__ void bar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void bar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// One tile (box fixed by the tensor map) from global to shared memory; completion is counted in bytes on `bar`.
+// x = innermost coordinate in elements (always 0 here), y = first row, z = first atom.
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, int32_t x, int32_t y, int32_t z, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+                 ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
+}
+// Asks for one tile of a tensor to be brought into L2 (no destination, no completion).
+__device__ __forceinline__ void tma_prefetch_3d(const CUtensorMap* tm, int32_t x, int32_t y, int32_t z) {
+    asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];"
+                 ::"l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(z) : "memory");
 }
 // Non-blocking test of an mbarrier phase.
 __device__ __forceinline__ bool bar_test(uint32_t bar, uint32_t parity) {
@@ -342,7 +357,8 @@ struct TcKernelParams {
 #endif
 };
 
-__global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams p) {
+__global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams p, const __grid_constant__ CUtensorMap tm_hi,
+                                                            const __grid_constant__ CUtensorMap tm_lo) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
     __shared__ uint32_t tmem_base_s;
@@ -358,14 +374,12 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
 
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SM_BAR);
     auto BAR = [&](int i) { return smem_u32(&bars[i]); };
-    float* sd_s = reinterpret_cast<float*>(smem + SM_SD);
-    float* kap_s = reinterpret_cast<float*>(smem + SM_KAP);
 
     if (tid == 0) {
         abort_s = 0;
         decision_s[0] = 0;
         decision_s[1] = 0;
-        bar_init(BAR(B_YFULL0), TR_THREADS);  bar_init(BAR(B_YFULL1), TR_THREADS);
+        bar_init(BAR(B_YFULL0), 1);    bar_init(BAR(B_YFULL1), 1);      // one arrive.expect_tx by the producer + the TMA bytes
         bar_init(BAR(B_YEMPTY0), 1);   bar_init(BAR(B_YEMPTY1), 1);
         bar_init(BAR(B_LFULL0), 1);    bar_init(BAR(B_LFULL1), 1);
         bar_init(BAR(B_RREADY0), 256); bar_init(BAR(B_RREADY1), 256);
@@ -377,7 +391,6 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(512) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    if (tid < 128) { sd_s[tid] = p.sd[tid]; kap_s[tid] = p.kap[tid]; }
     // P_lo image -> shared memory (plain 16-byte copies; the image is already swizzled)
     {
         const uint4* src = reinterpret_cast<const uint4*>(p.plo_img + (size_t)rank * 65536);
@@ -456,7 +469,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
             TIC(tk_);
             if (!bar_wait(BAR(B_LFULL0 + s), ph, abort_flag, p.status, false)) alive = false;
             TOC(tk_, 0);
-            if (gtid == 0) TRACE(0, i);
+            if (gtid == 0) TRACE(grp ? 14 : 0, i);
             fence_after();
 #ifdef FLASHGMM_DEBUG
             if (p.order & 4) {                // what-if timing only: no softmax work at all
@@ -687,7 +700,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
             fence_before();
             bar_arrive(BAR(B_RREADY0 + s));
             TOC(tk_, 7);
-            if (gtid == 0) TRACE(4, i);
+            if (gtid == 0) TRACE(grp ? 15 : 4, i);
             if (gtid < 32 && ll_have) {              // two-sum: (ll_s, ll_c) += log2 Z_i exactly to fp32 pair precision
                 const float v = ll_m + log2f(ll_z);
                 const float t = ll_s + v;
@@ -729,104 +742,67 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
             if (gtid == 0) {
                 double sum = 0.0;
                 for (int j = 0; j < 32; ++j) sum += lls[j];
-                p.llpart[cluster_id * 2 + grp] = sum * 0.69314718055994530942;
+                p.llpart[cluster_id * 2 + grp] += sum * 0.69314718055994530942;      // one owner per slot: launches add up
+            }
+        }
+    } else if (warp == PRODUCER_WARP) {
+        // =========================== producer warp: Y planes -> shared memory by TMA ===========================
+        // The fp16 planes of Y = [s x | (s x)^2 + kap] were written once for all CTAs by tc_transform_kernel; a stage is
+        // 2 planes x 4 atoms of (64 points x 128 bytes): one 3-D box per plane, and TMA's 128-byte swizzle produces exactly
+        // the K-major layout the MMA descriptors describe.  The whole warp runs the loop; lane 0 waits, one elected lane issues.
+        const int n_atoms = (p.n_ks + 3) >> 2;
+        const uint32_t stage_bytes = (uint32_t)n_atoms * 2u * 8192u;
+        int64_t issued = 0;
+        bool ok = true;
+        for (int64_t i = 0; i < ntl && ok; ++i) {
+            const int s = (int)(i & 1);
+            const uint32_t ph = (uint32_t)((i >> 1) & 1);
+            const int32_t row0 = (int32_t)((cluster_id + i * p.Q) * BN);
+            TIC(tt_);
+            if (i >= 2) {
+                uint32_t w = 1;
+                if (lane == 0) w = bar_wait(BAR(B_YEMPTY0 + s), ph ^ 1, abort_flag, p.status, false) ? 1u : 0u;
+                w = __shfl_sync(0xffffffffu, w, 0);
+                if (!w) { ok = false; break; }
+            }
+            TOC(tt_, 10);
+            if (tid == PRODUCER_WARP * 32) TRACE(5, i);
+            if (elect_one()) {
+                const uint32_t bar = BAR(B_YFULL0 + s);
+                const uint32_t dst = smem_u32(smem + SM_Y + s * SM_YSTAGE);
+#ifdef FLASHGMM_DEBUG
+                if (p.order & 8) bar_arrive(bar);          // what-if timing only: no loads, the stage keeps what it holds
+                else {
+#endif
+                bar_expect_tx(bar, stage_bytes);
+                tma_load_3d(dst, &tm_hi, 0, row0, 0, bar);                 // box = (128 bytes, 64 points, n_atoms atoms)
+                tma_load_3d(dst + SM_YLO, &tm_lo, 0, row0, 0, bar);
+#ifdef FLASHGMM_DEBUG
+                }
+#endif
+                // The planes were written by another kernel and are larger than L2: ask for the tile this CTA will load
+                // two steps from now (the next one is already in flight for the other stage); one CTA of the group asks
+                // for all, in turn.
+                if (i + 2 < ntl && (int)(i % p.CL) == (int)rank) {
+                    const int32_t rown = (int32_t)((cluster_id + (i + 2) * p.Q) * BN);
+                    tma_prefetch_3d(&tm_hi, 0, rown, 0);
+                    tma_prefetch_3d(&tm_lo, 0, rown, 0);
+                }
+            }
+            __syncwarp();
+            issued = i + 1;
+            TOC(tt_, 11);
+            if (tid == PRODUCER_WARP * 32) TRACE(6, i);
+        }
+        // On an abort the consumer may never wait for the last loads: they must have landed before the CTA may exit.
+        if (!ok || *abort_flag) {
+            for (int64_t i = (issued > 2 ? issued - 2 : 0); i < issued; ++i) {
+                if (lane == 0) bar_wait(BAR(B_YFULL0 + (int)(i & 1)), (uint32_t)((i >> 1) & 1), abort_flag, p.status, false);
+                __syncwarp();
             }
         }
     } else if (warp < MMA_WARP) {
-        // =========================== transform warps: X -> Y planes ===========================
-        // 224 threads share the 1024 (point, 8-dimension group) units of a tile: unit u = tau + 224 n, point u / 16,
-        // group u % 16 (16 consecutive threads read one row: coalesced 32-byte pieces).  A tile is loaded and converted
-        // into its four fp16 planes in registers BEFORE the wait for the stage, so that only the shared-memory stores
-        // sit between the release of a stage and its next use.
-        const int tau = tid - 256;
-        // a thread's eight dimensions never change (224 is a multiple of 16): their scales and shifts stay in registers
-        float sdr[8], kpr[8];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) { sdr[j] = sd_s[(tau & 15) * 8 + j]; kpr[j] = kap_s[(tau & 15) * 8 + j]; }
-        const bool vec_ok = (p.D % 4 == 0) && ((reinterpret_cast<uintptr_t>(p.X) & 15) == 0);
-        constexpr int NU = 5;                               // ceil(1024 / 224)
-        for (int64_t i = 0; i < ntl; ++i) {
-            const int s = (int)(i & 1);
-            const uint32_t ph = (uint32_t)((i >> 1) & 1);
-            const int64_t row_base = (cluster_id + i * p.Q) * BN;
-            unsigned char* yhi = smem + SM_Y + s * SM_YSTAGE;
-            unsigned char* ylo = yhi + SM_YLO;
-            float4 xa[NU], xb[NU];
-#pragma unroll
-            for (int n = 0; n < NU; ++n) {
-                const int u = tau + n * TR_THREADS;
-                const int pt = u >> 4, ks = u & 15, d0 = ks * 8;
-                const int64_t row = row_base + pt;
-                const bool row_ok = (u < 1024) && (row < p.n);
-                const float* xr = p.X + row * p.D;
-                if (row_ok && vec_ok && d0 + 8 <= p.D) {
-                    xa[n] = __ldg(reinterpret_cast<const float4*>(xr + d0));
-                    xb[n] = __ldg(reinterpret_cast<const float4*>(xr + d0 + 4));
-                } else {
-                    float x[8];
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) x[j] = (row_ok && d0 + j < p.D) ? __ldg(xr + d0 + j) : 0.f;
-                    xa[n] = make_float4(x[0], x[1], x[2], x[3]);
-                    xb[n] = make_float4(x[4], x[5], x[6], x[7]);
-                }
-            }
-            uint4 vxh[NU], vxl[NU], vqh[NU], vql[NU];
-#pragma unroll
-            for (int n = 0; n < NU; ++n) {
-                const float x[8] = {xa[n].x, xa[n].y, xa[n].z, xa[n].w, xb[n].x, xb[n].y, xb[n].z, xb[n].w};
-                uint32_t xh[4], xl[4], qh[4], ql[4];
-#pragma unroll
-                for (int j = 0; j < 8; j += 2) {
-                    float u0 = x[j] * sdr[j], u1 = x[j + 1] * sdr[j + 1];
-                    u0 = fminf(fmaxf(u0, -240.f), 240.f);
-                    u1 = fminf(fmaxf(u1, -240.f), 240.f);
-                    const float q0 = fmaf(u0, u0, kpr[j]), q1 = fmaf(u1, u1, kpr[j + 1]);
-                    const __half2 h = __floats2half2_rn(u0, u1);
-                    const float2 hf = __half22float2(h);
-                    const __half2 g2 = __floats2half2_rn(u0 - hf.x, u1 - hf.y);
-                    const __half2 sq = __floats2half2_rn(q0, q1);
-                    const float2 sf = __half22float2(sq);
-                    const __half2 t2 = __floats2half2_rn(q0 - sf.x, q1 - sf.y);
-                    xh[j / 2] = *reinterpret_cast<const uint32_t*>(&h);
-                    xl[j / 2] = *reinterpret_cast<const uint32_t*>(&g2);
-                    qh[j / 2] = *reinterpret_cast<const uint32_t*>(&sq);
-                    ql[j / 2] = *reinterpret_cast<const uint32_t*>(&t2);
-                }
-                vxh[n] = make_uint4(xh[0], xh[1], xh[2], xh[3]);
-                vxl[n] = make_uint4(xl[0], xl[1], xl[2], xl[3]);
-                vqh[n] = make_uint4(qh[0], qh[1], qh[2], qh[3]);
-                vql[n] = make_uint4(ql[0], ql[1], ql[2], ql[3]);
-            }
-            TIC(tt_);
-            if (i >= 2) {
-                if (!bar_wait(BAR(B_YEMPTY0 + s), ph ^ 1, abort_flag, p.status, false)) break;
-            }
-            TOC(tt_, 10);
-            if (tau == 0) TRACE(5, i);
-#ifdef FLASHGMM_DEBUG
-            if (!(p.order & 8))               // what-if timing only: no shared-memory stores
-#endif
-#pragma unroll
-            for (int n = 0; n < NU; ++n) {
-                const int u = tau + n * TR_THREADS;
-                if (u < 1024) {
-                    const int pt = u >> 4, ks = u & 15;
-                    // 16-byte chunk index in the point's 512-byte row: 2 ks (x) and 2 ks + 1 (x^2)
-                    const int atom = ks >> 2;
-                    const int cx = ((2 * (ks & 3)) ^ (pt & 7)) << 4;
-                    const int cq = ((2 * (ks & 3) + 1) ^ (pt & 7)) << 4;
-                    const int base = atom * 8192 + pt * 128;
-                    *reinterpret_cast<uint4*>(yhi + base + cx) = vxh[n];
-                    *reinterpret_cast<uint4*>(yhi + base + cq) = vqh[n];
-                    *reinterpret_cast<uint4*>(ylo + base + cx) = vxl[n];
-                    *reinterpret_cast<uint4*>(ylo + base + cq) = vql[n];
-                }
-            }
-            fence_async_smem();
-            bar_arrive(BAR(B_YFULL0 + s));
-            TOC(tt_, 11);
-            if (tau == 0) TRACE(6, i);
-        }
+        // warps 9-14 have no role in the tile loop (they copy P_lo in the prologue and meet the others at the end)
     } else {
         // =========================== MMA warp ===========================
         // The whole warp runs this loop convergently; lane 0 does the (bounded) waits and broadcasts their outcome, one
@@ -1036,6 +1012,58 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
 }
 
 // ---------------------------------------------------------------------------------------------------------------
+// X -> the two fp16 planes of Y, once per launch of the tile kernel (the CTAs of a group all read the same tiles, so
+// converting inside the tile kernel repeated this work in every CTA and took issue slots from the softmax warps).
+// Row i of a plane holds 256 halves: k-step ks (8 dimensions) occupies halves [16 ks, 16 ks + 8) = s x and
+// [16 ks + 8, 16 ks + 16) = (s x)^2 + kap, i.e. the column order of the E-step contraction.  One thread converts one
+// (point, k-step) unit and writes 32 contiguous bytes per plane; 16 consecutive threads write one 512-byte row.
+// Rows n .. rows_padded - 1 are written as zeros so that the last tile's loads need no out-of-bounds handling.
+__global__ void __launch_bounds__(256) tc_transform_kernel(const float* __restrict__ X, int64_t n, int64_t rows_padded, int D,
+                                                           const float* __restrict__ sd, const float* __restrict__ kap,
+                                                           unsigned char* __restrict__ yhi, unsigned char* __restrict__ ylo) {
+    const bool vec_ok = (D % 4 == 0) && ((reinterpret_cast<uintptr_t>(X) & 15) == 0);
+    const int64_t units = rows_padded * 16;
+    for (int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; u < units; u += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t row = u >> 4;
+        const int ks = (int)(u & 15), d0 = ks * 8;
+        float x[8];
+        if (row < n && vec_ok && d0 + 8 <= D) {
+            const float4 a = __ldg(reinterpret_cast<const float4*>(X + row * D + d0));
+            const float4 b = __ldg(reinterpret_cast<const float4*>(X + row * D + d0 + 4));
+            x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
+        } else {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) x[j] = (row < n && d0 + j < D) ? __ldg(X + row * D + d0 + j) : 0.f;
+        }
+        uint32_t xh[4], xl[4], qh[4], ql[4];
+#pragma unroll
+        for (int j = 0; j < 8; j += 2) {
+            float u0 = x[j] * __ldg(sd + d0 + j), u1 = x[j + 1] * __ldg(sd + d0 + j + 1);
+            u0 = fminf(fmaxf(u0, -240.f), 240.f);
+            u1 = fminf(fmaxf(u1, -240.f), 240.f);
+            float q0 = fmaf(u0, u0, __ldg(kap + d0 + j)), q1 = fmaf(u1, u1, __ldg(kap + d0 + j + 1));
+            if (row >= n) { q0 = 0.f; q1 = 0.f; }
+            const __half2 h = __floats2half2_rn(u0, u1);
+            const float2 hf = __half22float2(h);
+            const __half2 g2 = __floats2half2_rn(u0 - hf.x, u1 - hf.y);
+            const __half2 sq = __floats2half2_rn(q0, q1);
+            const float2 sf = __half22float2(sq);
+            const __half2 t2 = __floats2half2_rn(q0 - sf.x, q1 - sf.y);
+            xh[j / 2] = *reinterpret_cast<const uint32_t*>(&h);
+            xl[j / 2] = *reinterpret_cast<const uint32_t*>(&g2);
+            qh[j / 2] = *reinterpret_cast<const uint32_t*>(&sq);
+            ql[j / 2] = *reinterpret_cast<const uint32_t*>(&t2);
+        }
+        uint4* oh = reinterpret_cast<uint4*>(yhi + row * 512 + ks * 32);
+        uint4* ol = reinterpret_cast<uint4*>(ylo + row * 512 + ks * 32);
+        oh[0] = make_uint4(xh[0], xh[1], xh[2], xh[3]);
+        oh[1] = make_uint4(qh[0], qh[1], qh[2], qh[3]);
+        ol[0] = make_uint4(xl[0], xl[1], xl[2], xl[3]);
+        ol[1] = make_uint4(ql[0], ql[1], ql[2], ql[3]);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------------------
 // Parameter preparation for the tensor path (float64 arithmetic, K*D elements: negligible)
 
 // s_d = 2^-round(log2 rms_d) with rms_d^2 = sum_k pi_k (mu_kd^2 + var_kd): brings every dimension to O(1) so that the
@@ -1207,7 +1235,7 @@ extern "C" void gmm_debug_set_select(int cluster, int i) { g_tc_dbg_cluster = cl
 extern "C" void gmm_debug_set_clk(long long* p) { g_tc_clk = p; }
 #endif
 
-int g_tc_order = 1;
+int g_tc_order = 2;
 void tc_set_order(int o) { g_tc_order = o; }
 
 bool tc_supports(int D, int K) { return D >= 1 && D <= 128 && K >= 1 && K <= 1024; }
@@ -1232,6 +1260,7 @@ size_t tc_scratch_bytes(int D, int K) {
     b += (size_t)pl.Q * pl.Kpad * TC_PCOLS * 8;            // float64 partials
     b += (size_t)pl.Q * 16;
     b += 5 * (size_t)pl.Q * 4 * pl.CL * 64 * 16;           // exchange slots
+    b += 2 * TC_YPLANE_BYTES;                              // fp16 planes of Y for one launch
     return b + 8 * 256;
 }
 
@@ -1247,6 +1276,45 @@ cudaError_t launch_prepare_tc(cudaStream_t s, int D, int K, const float* pi, con
     tc_prepare_kernel<<<pl.Kpad, 128, 0, s>>>(D, K, pi, mu, var, tb.sd, tb.kap, tb.phi_img, tb.plo_img, tb.tk, tb.ck, tb.illb, cond_limit, tb.flags);
     return cudaGetLastError();
 }
+
+cudaError_t launch_transform_tc(cudaStream_t s, const float* X, int64_t n, int D, const TcBuffers& tb) {
+    if (n < 1 || n > TC_YPOINTS) return cudaErrorInvalidValue;
+    const int64_t rows_padded = (n + TC_BN - 1) / TC_BN * TC_BN;
+    const int64_t units = rows_padded * 16;
+    int64_t blocks = (units + 255) / 256;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    tc_transform_kernel<<<(unsigned)blocks, 256, 0, s>>>(X, n, rows_padded, D, tb.sd, tb.kap, tb.y_hi, tb.y_lo);
+    return cudaGetLastError();
+}
+
+namespace {
+// A plane [rows][256 halves] seen as a 3-D tensor (x = 64 halves of an atom's row, y = row, z = atom): a box of
+// (64, 64 points, n_atoms) lands in shared memory as [atom][point][128 bytes], each 128-byte row swizzled.
+cudaError_t make_plane_map(CUtensorMap* tm, void* base, int64_t rows, int n_atoms) {
+    const cuuint64_t dims[3] = {64, (cuuint64_t)rows, 4};
+    const cuuint64_t strides[2] = {512, 128};                 // bytes between rows, between atoms
+    const cuuint32_t box[3] = {64, (cuuint32_t)TC_BN, (cuuint32_t)n_atoms};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    // The encoder lives in the driver library; it is looked up at run time so that this library has no load-time
+    // dependency on the driver (it must load, e.g. for symbol checks, on a machine without one).
+    typedef CUresult (*encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    static encode_fn encode = nullptr;
+    if (!encode) {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        const cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
+        if (e != cudaSuccess) return e;
+        if (q != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
+        encode = reinterpret_cast<encode_fn>(fn);
+    }
+    const CUresult r = encode(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, base, dims, strides, box, estr,
+                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+}  // namespace
 
 cudaError_t launch_em_tc(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu, const float* w2,
                          const float* c2, const TcBuffers& tb, int Q, int flush_tiles, int* status) {
@@ -1285,7 +1353,15 @@ cudaError_t launch_em_tc(cudaStream_t s, const float* X, int64_t n, int D, int K
     attr[0].val.cooperative = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, em_tc_kernel, p);
+    if (n < 1 || n > TC_YPOINTS) return cudaErrorInvalidValue;
+    const int64_t rows_padded = (n + TC_BN - 1) / TC_BN * TC_BN;       // launch_transform_tc wrote zeros beyond n
+    CUtensorMap tm_hi, tm_lo;
+    const int n_atoms = (pl.n_ks + 3) / 4;
+    e = make_plane_map(&tm_hi, tb.y_hi, rows_padded, n_atoms);
+    if (e != cudaSuccess) return e;
+    e = make_plane_map(&tm_lo, tb.y_lo, rows_padded, n_atoms);
+    if (e != cudaSuccess) return e;
+    return cudaLaunchKernelEx(&cfg, em_tc_kernel, p, tm_hi, tm_lo);
 }
 
 // Number of groups (of ceil(K/128) CTAs, one CTA per SM) that can be resident at once: the persistent grid size.

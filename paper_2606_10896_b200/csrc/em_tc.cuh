@@ -10,6 +10,8 @@ constexpr int TC_BN = 64;            // points per tile
 constexpr int TC_FLUSH = 64;         // tiles between flushes of the TMEM accumulators into float64 partials (even)
 constexpr float TC_RSCALE = 4096.f;  // responsibilities are scaled by this power of two before the fp16 split
 constexpr int TC_PCOLS = 258;        // columns of a partial row: 256 statistics columns + N_k of each softmax group
+constexpr int64_t TC_YPOINTS = 1 << 19;   // points per launch of the tile kernel: capacity of the fp16 planes of Y in scratch
+constexpr size_t TC_YPLANE_BYTES = (size_t)TC_YPOINTS * 512;   // one plane: 256 fp16 values per point
 
 struct TcPlan {
     int CL;     // CTAs per group = ceil(K / 128)
@@ -31,15 +33,20 @@ struct TcBuffers {
     double* llpart;
     void* xg;   // exchange slots of the log-sum-exp, [Q][4][CL][64] x 16 bytes
     void* xl;   // exchange slots of the lower-bound pass
+    unsigned char* y_hi;   // [TC_YPOINTS][256] fp16: high parts of Y = [s x | (s x)^2 + kap], k-step interleaved
+    unsigned char* y_lo;   // the low parts
 };
 
 bool tc_supports(int D, int K);
-void tc_set_order(int o);   // MMA issue order: 0 = pairs E E M M, 1 = interleaved M(i) E(i+2) (default), 2 = whichever of E(i+2), M(i+1) is ready first
+void tc_set_order(int o);   // MMA issue order: 0 = pairs E E M M, 1 = interleaved M(i) E(i+2), 2 = whichever of E(i+2), M(i+1) is ready first (default)
 TcPlan tc_plan(int D, int K, int num_sms);
 size_t tc_scratch_bytes(int D, int K);
 cudaError_t tc_max_clusters(int D, int K, int* out);
 cudaError_t launch_prepare_tc(cudaStream_t s, int D, int K, const float* pi, const float* mu, const float* var,
                               const TcBuffers& tb, float cond_limit, int* status);
+// One pass over at most TC_YPOINTS points: X -> the two fp16 planes of Y in scratch (read by the tile kernel through TMA).
+cudaError_t launch_transform_tc(cudaStream_t s, const float* X, int64_t n, int D, const TcBuffers& tb);
+// n <= TC_YPOINTS points whose planes launch_transform_tc has written.
 // mu, w2, c2: the FP32 path's derived parameters (launch_prepare_fp32), used to recompute ill-conditioned logits exactly
 cudaError_t launch_em_tc(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu, const float* w2,
                          const float* c2, const TcBuffers& tb, int Q, int flush_tiles, int* status);

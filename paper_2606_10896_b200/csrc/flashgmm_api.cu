@@ -28,11 +28,12 @@ inline size_t align256(size_t b) { return (b + 255) & ~(size_t)255; }
 
 struct ScratchLayout {
     size_t w2, c2, c2d, partials, logZ2, llpart, result, stats, total;
-    size_t tc_phi, tc_plo, tc_tk, tc_ck, tc_sd, tc_kap, tc_illb, tc_flags, tc_xg, tc_xl, tc_partial, tc_llpart, tc_partial_bytes;
+    size_t tc_phi, tc_plo, tc_tk, tc_ck, tc_sd, tc_kap, tc_illb, tc_flags, tc_xg, tc_xl, tc_partial, tc_llpart, tc_partial_bytes, tc_yhi, tc_ylo;
     bool tc;
 };
 
-ScratchLayout scratch_layout(int D, int K) {
+// planes: include the fp16 planes of Y (tensor path only; 2 x TC_YPLANE_BYTES, placed last so that no other offset moves)
+ScratchLayout scratch_layout(int D, int K, bool planes) {
     ScratchLayout L;
     const size_t KD = (size_t)K * D;
     size_t off = 0;
@@ -46,7 +47,7 @@ ScratchLayout scratch_layout(int D, int K) {
     L.result = take(sizeof(DevResult));
     L.stats = take(((size_t)K + 2 * KD) * 8);
     L.tc = tc_supports(D, K);
-    L.tc_phi = L.tc_plo = L.tc_tk = L.tc_ck = L.tc_sd = L.tc_kap = L.tc_illb = L.tc_flags = L.tc_xg = L.tc_xl = L.tc_partial = L.tc_llpart = 0;
+    L.tc_phi = L.tc_plo = L.tc_tk = L.tc_ck = L.tc_sd = L.tc_kap = L.tc_illb = L.tc_flags = L.tc_xg = L.tc_xl = L.tc_partial = L.tc_llpart = L.tc_yhi = L.tc_ylo = 0;
     L.tc_partial_bytes = 0;
     if (L.tc) {
         const TcPlan pl = tc_plan(D, K, 160);       // an upper bound on the number of clusters
@@ -64,6 +65,10 @@ ScratchLayout scratch_layout(int D, int K) {
         L.tc_partial = take(L.tc_partial_bytes);
         L.tc_llpart = take((size_t)pl.Q * 16);
     }
+    if (L.tc && planes) {
+        L.tc_yhi = take(TC_YPLANE_BYTES);
+        L.tc_ylo = take(TC_YPLANE_BYTES);
+    }
     L.total = off;
     return L;
 }
@@ -80,11 +85,13 @@ struct gmm_ctx {
     unsigned char* scratch = nullptr;
     size_t scratch_bytes = 0;
     int capD = 0, capK = 0;
+    bool capPlanes = false;    // the scratch layout in force includes the tensor path's planes of Y
     ScratchLayout lay{};
     int tc_Q = 0;              // resident clusters of the tensor-path kernel for (capD, capK)
     float tc_cond_limit = -1.f;      // < 0: automatic, tc_cond_scale * sqrt(N / K)
     float tc_cond_scale = 1.5e-4f;
     int tc_flush = TC_FLUSH;
+    int64_t tc_piece = TC_YPOINTS;   // points per launch of the tile kernel (<= capacity of the Y planes)
     // host-streaming path
     cudaStream_t copy_stream = nullptr;
     float* xstage[2] = {nullptr, nullptr};
@@ -123,6 +130,8 @@ struct gmm_ctx {
         b.xl = scratch + lay.tc_xl;
         b.partial = reinterpret_cast<double*>(scratch + lay.tc_partial);
         b.llpart = reinterpret_cast<double*>(scratch + lay.tc_llpart);
+        b.y_hi = scratch + lay.tc_yhi;
+        b.y_lo = scratch + lay.tc_ylo;
         return b;
     }
 };
@@ -154,9 +163,13 @@ int fail(gmm_ctx* ctx, int code, const char* fmt, ...) {
         ctx->launches++;                                                                              \
     } while (0)
 
+// The tensor path runs when it is forced or when AUTO picks it for the shape: only then are the planes of Y needed.
+bool auto_is_tensor(int D, int K) { return tc_supports(D, K) && K >= 64 && D >= 8; }
+
 int ensure_scratch(gmm_ctx* ctx, int D, int K) {
-    if (ctx->scratch && D == ctx->capD && K == ctx->capK) return GMM_OK;
-    const ScratchLayout L = scratch_layout(D, K);
+    const bool planes = tc_supports(D, K) && (ctx->path == GMM_PATH_TENSOR || (ctx->path == GMM_PATH_AUTO && auto_is_tensor(D, K)));
+    if (ctx->scratch && D == ctx->capD && K == ctx->capK && planes == ctx->capPlanes) return GMM_OK;
+    const ScratchLayout L = scratch_layout(D, K, planes);
     if (L.total > ctx->scratch_bytes) {
         if (ctx->scratch) {
             CU(cudaStreamSynchronize(ctx->stream));
@@ -176,6 +189,7 @@ int ensure_scratch(gmm_ctx* ctx, int D, int K) {
     ctx->lay = L;
     ctx->capD = D;
     ctx->capK = K;
+    ctx->capPlanes = planes;
     ctx->tc_Q = 0;
     if (L.tc) {
         int q = 0;
@@ -270,9 +284,16 @@ int accumulate_points(gmm_ctx* ctx, int path, const float* X, int64_t n, int D, 
         const int Q = ctx->tc_Q;
         CU(cudaMemsetAsync(tb.partial, 0, (size_t)Q * pl.Kpad * TC_PCOLS * 8, ctx->stream));
         CU(cudaMemsetAsync(tb.llpart, 0, (size_t)Q * 16, ctx->stream));
-        CHECK(prof_begin(ctx));
-        KL(launch_em_tc(ctx->stream, X, n, D, K, mu, ctx->w2(), ctx->c2(), tb, Q, ctx->tc_flush, &ctx->result()->status));
-        CHECK(prof_end(ctx));
+        // The fp16 planes of Y are built once per launch-sized piece of X (not once per CTA of a group), so the tile kernel
+        // is launched per piece; its float64 partials and log-likelihood partials accumulate across the launches.
+        for (int64_t off = 0; off < n; off += ctx->tc_piece) {
+            const int64_t cnt = (n - off < ctx->tc_piece) ? (n - off) : ctx->tc_piece;
+            const float* Xs = X + off * D;
+            CHECK(prof_begin(ctx));
+            KL(launch_transform_tc(ctx->stream, Xs, cnt, D, tb));
+            KL(launch_em_tc(ctx->stream, Xs, cnt, D, K, mu, ctx->w2(), ctx->c2(), tb, Q, ctx->tc_flush, &ctx->result()->status));
+            CHECK(prof_end(ctx));
+        }
         KL(launch_reduce_ll(ctx->stream, tb.llpart, 2 * Q, &ctx->result()->ll[slot], true));
         KL(launch_reduce_tc(ctx->stream, D, K, Q, tb, Nk, S1, S2, true));
         return GMM_OK;
@@ -344,9 +365,13 @@ int gmm_create(gmm_ctx** out, int device, void* cuda_stream) {
     ctx->stream = static_cast<cudaStream_t>(cuda_stream);
     if (const char* e = std::getenv("GMM_TC_COND_LIMIT")) ctx->tc_cond_limit = (float)std::atof(e);
     if (const char* e = std::getenv("GMM_TC_FLUSH")) ctx->tc_flush = std::atoi(e);
+    if (const char* e = std::getenv("GMM_TC_PIECE")) {
+        const long long v = std::atoll(e);
+        if (v >= 64 && v <= TC_YPOINTS) ctx->tc_piece = v / 64 * 64;
+    }
     {   // the issue order is process-wide: every create sets it, so a context never inherits an earlier context's choice
         const char* e = std::getenv("GMM_TC_ORDER");
-        tc_set_order(e ? std::atoi(e) : 1);
+        tc_set_order(e ? std::atoi(e) : 2);
     }
     *out = ctx;
     return GMM_OK;
@@ -586,11 +611,11 @@ int gmm_assign_topm(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const
 
 int gmm_tensor_path_supports(int D, int K) { return tc_supports(D, K) ? 1 : 0; }
 
-int gmm_auto_path(int D, int K) { return (tc_supports(D, K) && K >= 64 && D >= 8) ? GMM_PATH_TENSOR : GMM_PATH_FP32; }
+int gmm_auto_path(int D, int K) { return auto_is_tensor(D, K) ? GMM_PATH_TENSOR : GMM_PATH_FP32; }
 
 size_t gmm_scratch_bytes(int D, int K) {
     if (D < 1 || K < 1) return 0;
-    return scratch_layout(D, K).total;
+    return scratch_layout(D, K, auto_is_tensor(D, K)).total;      // what a context in GMM_PATH_AUTO allocates
 }
 
 int64_t gmm_launch_count(const gmm_ctx* ctx) { return ctx ? ctx->launches : 0; }

@@ -16,14 +16,15 @@
 //
 // Layout: lanes of TMEM = components.  TMEM columns: [0,256) statistics accumulator, [256,384) P_hi (fp16 pairs),
 // [384,448) / [448,512) logits of the two tiles in flight (overwritten in place by r_hi | r_lo).
-// Shared memory: P_lo (64 KB, SW128 K-major), two stages of Y (hi and lo planes, SW128; read K-major by the E-step and
-// MN-major by the M-step), exchange buffers, barriers.
+// Shared memory: P_lo (64 KB, SW128 K-major), two stages of Y (hi and lo planes, written by TMA with the 128-byte swizzle;
+// read K-major by the E-step and MN-major by the M-step), exchange buffers, barriers.
 //
-// Warp roles: warps 0-7 softmax (two warpgroups, each taking 32 of a tile's 64 points; warp w owns TMEM lanes
-// 32 (w mod 4) ...), warps 8-14 load X with coalesced 16-byte loads and build the Y planes, warp 15 issues the MMAs: the
-// whole warp runs the issue loop convergently, lane 0 does the waits and broadcasts their outcome, one elected lane
-// issues (descriptors = hoisted base + immediate offset, loops unrolled) and commits.  Three issue orders exist (pairs,
-// interleaved = default, whichever-is-ready); all give identical results.  Every wait is bounded by a wall-clock limit;
+// Warp roles (10 warps): warps 0-7 softmax (two warpgroups, each taking 32 of a tile's 64 points; warp w owns TMEM lanes
+// 32 (w mod 4) ...), warp 8 produces the Y stages (TMA loads of the fp16 planes that tc_transform_kernel wrote once for
+// all CTAs, one 3-D box per plane, L2 prefetch two tiles ahead), warp 9 issues the MMAs: the whole warp runs the issue loop
+// convergently, lane 0 does the waits and broadcasts their outcome, one elected lane issues (descriptors = hoisted base +
+// immediate offset, loops unrolled) and commits.  Three issue orders exist (pairs, interleaved, whichever-is-ready =
+// default); all give identical results.  Every wait is bounded by a wall-clock limit;
 // on expiry the CTA sets ST_TIMEOUT, all roles leave their loops, TMEM is freed and the kernel returns.
 #include "internal.cuh"
 #include "em_tc.cuh"
@@ -40,8 +41,8 @@ namespace fg {
 namespace {
 
 constexpr int BN = TC_BN;                 // points per tile
-constexpr int NTHREADS = 512;          // 8 softmax warps, 7 transform warps, 1 MMA warp (16 warps: 128 registers each)
-constexpr int MMA_WARP = 15;
+constexpr int NTHREADS = 320;          // 8 softmax warps, 1 producer warp, 1 MMA warp (10 warps: up to 200 registers each)
+constexpr int MMA_WARP = 9;
 constexpr int PRODUCER_WARP = 8;
 constexpr float RSCALE = TC_RSCALE;
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
@@ -801,8 +802,6 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                 __syncwarp();
             }
         }
-    } else if (warp < MMA_WARP) {
-        // warps 9-14 have no role in the tile loop (they copy P_lo in the prologue and meet the others at the end)
     } else {
         // =========================== MMA warp ===========================
         // The whole warp runs this loop convergently; lane 0 does the (bounded) waits and broadcasts their outcome, one

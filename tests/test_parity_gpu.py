@@ -116,6 +116,16 @@ def test_tensor_ill_conditioned_mode_under_both_issue_orders(fg, order, monkeypa
         _teacher_forced(fg, c, synth.sample_host(spec), spec, 3, paths=[fg.GMM_PATH_TENSOR])
 
 
+def test_tensor_path_accumulates_over_pieces(fg, monkeypatch):
+    # The tensor path converts X to its fp16 planes and launches the tile kernel once per piece of points (2^19 by
+    # default).  With pieces of 1024 points a 3000-point problem takes three launches, the last one ragged (952 points,
+    # 14 tiles + a tail of 56): statistics and log-likelihood must still be those of one pass over all points.
+    monkeypatch.setenv("GMM_TC_PIECE", "1024")
+    spec = synth.CONFIGS[2].with_n(3000)
+    with fg.Context(0) as c:
+        _teacher_forced(fg, c, synth.sample_host(spec), spec, 2, paths=[fg.GMM_PATH_TENSOR])
+
+
 def test_config2_free_running_30_iterations(fg, ctx):
     """Config 2 as specified (N = 100,000, D = 128, K = 1024, 30 iterations): both sides iterate freely from the same
     initial parameters; the log-likelihood traces agree to 1e-4 relative at every iteration."""

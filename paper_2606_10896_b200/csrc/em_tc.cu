@@ -542,53 +542,103 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                     const int kglob = (int)rank * 128 + kloc;
                     bool fixed_any = false;
                     TOC(tk_, 29);
-                    for (;;) {
+                    // Second filter, against the GROUP-wide lower bound of each point (the maximum of the bounds that all
+                    // 4 CL warps of the group published).  That bound depends on the point only, so it is fetched once per
+                    // point that has candidates - four points per L2 round trip, lane c reading the slot of
+                    // (CTA c / 4, warp c % 4) - and not once per candidate pair: with half of the components flagged
+                    // (small N / K) two thousand pairs per tile pass the warp-local filter and a handful survive this one.
+                    // (at large N / K almost no tile has a candidate at all: one ballot decides, and the rest is skipped)
+                    const bool have_cand = __ballot_sync(0xffffffffu, mlo != 0u) != 0u;
+                    uint32_t pm = have_cand ? __reduce_or_sync(0xffffffffu, mlo) : 0u;       // points with at least one candidate
+                    float lb_keep = CUDART_INF_F;                            // lane j keeps the group bound of point j
+                    while (pm != 0u && alive) {
+#ifdef FLASHGMM_DEBUG
+                        if (p.dbg_clk && blockIdx.x == 0 && lane == 0) atomicAdd((unsigned long long*)&p.dbg_clk[24], 1ull);
+                        if (p.dbg_clk && blockIdx.x == 0 && lane == 0) atomicAdd((unsigned long long*)&p.dbg_clk[23], (unsigned long long)__popc(pm));
+#endif
+                        int jb[4];
+                        uint32_t rest = pm;
+#pragma unroll
+                        for (int b8 = 0; b8 < 4; ++b8) {
+                            jb[b8] = rest ? (__ffs(rest) - 1) : -1;
+                            if (rest) rest &= rest - 1;
+                        }
+                        float lbv[4];
+                        unsigned long long t0 = 0;
+                        for (int it = 0;; ++it) {
+                            bool ok = true;
+#pragma unroll
+                            for (int b8 = 0; b8 < 4; ++b8) {
+                                lbv[b8] = -CUDART_INF_F;
+                                if (jb[b8] >= 0 && lane < 4 * p.CL) {
+                                    uint32_t v[4];
+                                    xslot_load(ring + lane * 64 + jb[b8], v);
+                                    if (v[1] == tag && v[3] == tag) lbv[b8] = __uint_as_float(v[0]);
+                                    else ok = false;
+                                }
+                            }
+                            if (__all_sync(0xffffffffu, ok)) break;
+                            bool give_up = *abort_flag != 0;
+                            if ((it & 15) == 15) {
+                                const unsigned long long now = gtime();
+                                if (t0 == 0) t0 = now;
+                                else if (now - t0 > WAIT_LIMIT_NS) {
+                                    *abort_flag = 1;
+                                    atomicOr(p.status, ST_TIMEOUT);
+                                    give_up = true;
+                                }
+                            }
+                            if (__any_sync(0xffffffffu, give_up)) { alive = false; break; }
+                        }
+                        if (!alive) break;
+#pragma unroll
+                        for (int b8 = 0; b8 < 4; ++b8) {
+                            if (jb[b8] < 0) continue;                       // uniform: jb is the same in every lane
+                            float m = lbv[b8];
+#pragma unroll
+                            for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+                            if (lane == jb[b8]) lb_keep = m;
+                        }
+                        pm = rest;
+                    }
+                    if (have_cand && alive) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const float lbj = __shfl_sync(0xffffffffu, lb_keep, j);
+                            if (((mlo >> j) & 1u) && !(l[j] + illb >= lbj - ILL_MARGIN)) mlo &= ~(1u << j);
+                        }
+                    } else {
+                        mlo = 0u;
+                    }
+                    // The survivors are recomputed exactly with direct differences in fp32, the whole warp on one pair.
+                    while (have_cand) {
                         const uint32_t ballot = __ballot_sync(0xffffffffu, mlo != 0u);
                         if (ballot == 0u) break;
                         const int src = __ffs(ballot) - 1;
                         int j = __ffs(mlo) - 1;
-                        float ub = -CUDART_INF_F;                  // upper bound l + E of the owner's candidate
+                        j = __shfl_sync(0xffffffffu, j, src);
+                        const int kk = __shfl_sync(0xffffffffu, kglob, src);
+#ifdef FLASHGMM_DEBUG
+                        if (p.dbg_clk && blockIdx.x == 0 && lane == 0) atomicAdd((unsigned long long*)&p.dbg_clk[25], 1ull);
+#endif
+                        const float* xr = p.X + (row0 + p0 + j) * p.D;
+                        const float* mr = p.mu + (size_t)kk * p.D;
+                        const float* wr = p.w2 + (size_t)kk * p.D;
+                        float q = 0.f;
+                        for (int d = lane; d < p.D; d += 32) {
+                            const float diff = __ldg(xr + d) - __ldg(mr + d);
+                            q = fmaf(diff * diff, __ldg(wr + d), q);
+                        }
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
+                        const float val = __ldg(p.c2 + kk) - q;
                         if (lane == src) {
 #pragma unroll
                             for (int jj = 0; jj < 32; ++jj)
-                                if (jj == j) ub = l[jj] + illb;
+                                if (jj == j) l[jj] = val;
+                            mlo &= ~(1u << j);
                         }
-                        j = __shfl_sync(0xffffffffu, j, src);
-                        ub = __shfl_sync(0xffffffffu, ub, src);
-                        const int kk = __shfl_sync(0xffffffffu, kglob, src);
-                        // group-wide lower-bound maximum of point j: lane c reads the slot of (CTA c / 4, warp c % 4)
-                        float lbv = -CUDART_INF_F, dummy = 0.f;
-                        if (lane < 4 * p.CL) {
-                            if (!xslot_wait(ring + lane * 64 + j, tag, lbv, dummy, abort_flag, p.status)) alive = false;
-                        }
-#pragma unroll
-                        for (int o = 16; o > 0; o >>= 1) lbv = fmaxf(lbv, __shfl_xor_sync(0xffffffffu, lbv, o));
-#ifdef FLASHGMM_DEBUG
-                        if (p.dbg_clk && blockIdx.x == 0 && lane == 0) atomicAdd((unsigned long long*)&p.dbg_clk[24], 1ull);
-#endif
-                        if (ub >= lbv - ILL_MARGIN) {
-#ifdef FLASHGMM_DEBUG
-                            if (p.dbg_clk && blockIdx.x == 0 && lane == 0) atomicAdd((unsigned long long*)&p.dbg_clk[25], 1ull);
-#endif
-                            const float* xr = p.X + (row0 + p0 + j) * p.D;
-                            const float* mr = p.mu + (size_t)kk * p.D;
-                            const float* wr = p.w2 + (size_t)kk * p.D;
-                            float q = 0.f;
-                            for (int d = lane; d < p.D; d += 32) {
-                                const float diff = __ldg(xr + d) - __ldg(mr + d);
-                                q = fmaf(diff * diff, __ldg(wr + d), q);
-                            }
-#pragma unroll
-                            for (int o = 16; o > 0; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
-                            const float val = __ldg(p.c2 + kk) - q;
-                            if (lane == src) {
-#pragma unroll
-                                for (int jj = 0; jj < 32; ++jj)
-                                    if (jj == j) l[jj] = val;
-                            }
-                            fixed_any = true;
-                        }
-                        if (lane == src) mlo &= ~(1u << j);
+                        fixed_any = true;
                     }
                     __syncwarp();
                     TOC(tk_, 30);

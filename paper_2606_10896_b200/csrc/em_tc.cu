@@ -57,11 +57,7 @@ constexpr int SM_MISC = SM_Y + 2 * SM_YSTAGE;   // 196608
 constexpr int SM_GATHER = SM_MISC;              // 2 groups x 4 warps x 64 floats    2048
 constexpr int SM_WS = SM_GATHER + 2048;         // 2 groups x 4 warps x 64 float2    4096
 constexpr int SM_FAC = SM_WS + 4096;            // 2 groups x 4 warps x 64 floats    2048
-constexpr int SM_LBW = SM_FAC + 2048;           // 2 groups x 4 warps x 64 floats    2048
-constexpr int SM_LBG = SM_LBW + 2048;           // 2 groups x 64 floats               512
-constexpr int SM_SD = SM_LBG + 512;             // 128 floats                     512
-constexpr int SM_KAP = SM_SD + 512;             // 128 floats                     512
-constexpr int SM_LL = SM_KAP + 512;             // 2 x 64 doubles                1024
+constexpr int SM_LL = SM_FAC + 2048;            // 2 x 64 doubles                1024
 constexpr int SM_BAR = SM_LL + 1024;             // barriers                       256
 constexpr int SM_END = SM_BAR + 256;
 constexpr int SMEM_BYTES = SM_END + 1024;       // + alignment slack
@@ -200,26 +196,6 @@ __device__ __forceinline__ bool bar_wait(uint32_t bar, uint32_t parity, volatile
     }
 }
 
-// Bounded poll of an exchange slot until both tags match.
-__device__ __forceinline__ bool xslot_wait(const XSlot* q, uint32_t tag, float& a, float& b, volatile int* abort_flag, int* status) {
-    unsigned long long t0 = 0;
-    for (int it = 0;; ++it) {
-        uint32_t v[4];
-        xslot_load(q, v);
-        if (v[1] == tag && v[3] == tag) { a = __uint_as_float(v[0]); b = __uint_as_float(v[2]); return true; }
-        if (*abort_flag) return false;
-        if ((it & 63) == 63) {
-            const unsigned long long now = gtime();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > WAIT_LIMIT_NS) {
-                *abort_flag = 1;
-                atomicOr(status, ST_TIMEOUT);
-                return false;
-            }
-        }
-    }
-}
-
 // Bounded poll of the CL slots of one point (stride 64 slots between source CTAs): all outstanding loads are issued
 // together, so one round costs one L2 round trip.  Called by a whole warp, one point per lane; the warp leaves the loop
 // TOGETHER (when every lane has all its slots): lanes that left at different rounds would run the code that follows
@@ -325,9 +301,6 @@ __device__ __forceinline__ void warp_reduce_scatter32(const float (&v)[32], floa
     out = e[0];
 }
 
-__device__ __forceinline__ uint32_t pack_h2(__half lo, __half hi) {
-    return (uint32_t)__half_as_ushort(lo) | ((uint32_t)__half_as_ushort(hi) << 16);
-}
 
 struct TcKernelParams {
     const float* X;
@@ -337,8 +310,6 @@ struct TcKernelParams {
     const unsigned char* plo_img;  // [CL][65536] shared-memory image (SW128, K-major)
     const float* tk;               // [CL*128]
     const float* ck;               // [CL*128]
-    const float* sd;               // [128] per-dimension power-of-two data scale
-    const float* kap;              // [128] per-dimension shift of the squares: Y = [s x | (s x)^2 + kap]
     const float* illb;             // [CL*128] 0, or for an ill-conditioned component a bound E_k on the error of its approximate log2 z
     const int* flags;              // [0] != 0 when some component is ill-conditioned (kernel-uniform protocol switch)
     const float* mu;               // [K][D] means (exact recomputation)
@@ -1372,7 +1343,7 @@ cudaError_t launch_em_tc(cudaStream_t s, const float* X, int64_t n, int D, int K
     p.X = X; p.n = n; p.D = D; p.K = K; p.CL = pl.CL; p.Q = Q; p.n_ks = pl.n_ks;
     p.flush = (flush_tiles < 2) ? 2 : (flush_tiles & ~1);
     p.order = g_tc_order;
-    p.phi_img = tb.phi_img; p.plo_img = tb.plo_img; p.tk = tb.tk; p.ck = tb.ck; p.sd = tb.sd; p.kap = tb.kap;
+    p.phi_img = tb.phi_img; p.plo_img = tb.plo_img; p.tk = tb.tk; p.ck = tb.ck;
     p.illb = tb.illb; p.flags = tb.flags; p.mu = mu; p.w2 = w2; p.c2 = c2;
     p.partial = tb.partial; p.llpart = tb.llpart; p.status = status;
     p.xg = static_cast<XSlot*>(tb.xg); p.xl = static_cast<XSlot*>(tb.xl);

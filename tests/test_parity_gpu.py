@@ -142,7 +142,7 @@ def test_config2_free_running_30_iterations(fg, ctx):
 
 
 @pytest.mark.parametrize("N,D,K", [(1, 1, 1), (127, 16, 8), (129, 96, 129), (64, 100, 1), (1000, 3, 65),
-                                    (257, 128, 128), (333, 130, 70)])
+                                    (257, 128, 128), (333, 130, 70), (500, 100, 200), (300, 30, 64), (700, 9, 1000)])
 def test_odd_shapes_one_step(fg, ctx, N, D, K):
     rng = np.random.Generator(np.random.PCG64(N * 1000 + D * 10 + K))
     mu = rng.normal(0, 2, (K, D))
@@ -157,6 +157,29 @@ def test_odd_shapes_one_step(fg, ctx, N, D, K):
         got = _gpu_step(ctx, _t(X), p32, m32, v32)
         assert abs(got[3] - ref[3]) <= 1e-5 * abs(ref[3]) + 1e-6
         assert_stats_close(N, s, got[:3], ref[:3], f"path {path} shape {(N, D, K)}")
+
+
+def test_x_pointer_that_is_only_4_byte_aligned(fg, ctx):
+    # Both paths use 16-byte loads of X when they can; a view that starts one float into an allocation must take the scalar
+    # loads and give the same statistics.
+    N, D, K = 333, 96, 129
+    rng = np.random.Generator(np.random.PCG64(7))
+    mu = rng.normal(0, 2, (K, D))
+    var = rng.uniform(0.3, 2.0, (K, D))
+    pi = rng.dirichlet(np.ones(K))
+    X = (mu[rng.integers(0, K, N)] + rng.standard_normal((N, D))).astype(np.float32)
+    s = max(data_scale(X), 1.0)
+    p32, m32, v32 = pi.astype(np.float32), mu.astype(np.float32), var.astype(np.float32)
+    ref = orc.em_step(X, p32, m32, v32)
+    buf = torch.empty(N * D + 1, dtype=torch.float32, device=DEV)
+    X_d = buf[1:].view(N, D)
+    X_d.copy_(torch.from_numpy(X))
+    assert X_d.data_ptr() % 16 == 4
+    for path in _paths(fg, D, K):
+        ctx.gmm_set_path(path)
+        got = _gpu_step(ctx, X_d, p32, m32, v32)
+        assert abs(got[3] - ref[3]) <= 1e-5 * abs(ref[3]) + 1e-6
+        assert_stats_close(N, s, got[:3], ref[:3], f"path {path}, X misaligned")
 
 
 @pytest.mark.parametrize("N,D,K", [(1, 1, 1), (127, 16, 8), (64, 100, 1), (333, 60, 33)])

@@ -45,7 +45,9 @@ constexpr int NTHREADS = 320;          // 8 softmax warps, 1 producer warp, 1 MM
 constexpr int MMA_WARP = 9;
 constexpr int PRODUCER_WARP = 8;
 constexpr float RSCALE = TC_RSCALE;
-constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
+// Wall-clock limit of every device-side wait, in ns (2 s; a test of the time-out path shortens it).
+__constant__ unsigned long long c_wait_limit_ns = 2000000000ull;
+#define WAIT_LIMIT_NS c_wait_limit_ns
 constexpr float ILL_MARGIN = 40.f;     // log2 units: a logit more than this below the best one is negligible (2^-40)
 
 // shared memory map (offsets from a 1024-byte aligned base)
@@ -306,6 +308,7 @@ struct TcKernelParams {
     const float* X;
     int64_t n;
     int D, K, CL, Q, n_ks, flush, order;
+    int test_silent_rank;          // >= 0: that CTA of group 0 never publishes its exchange slot for tile 0 (time-out test)
     const uint32_t* phi_img;       // [CL][128 lanes][128] packed fp16 pairs
     const unsigned char* plo_img;  // [CL][65536] shared-memory image (SW128, K-major)
     const float* tk;               // [CL*128]
@@ -335,8 +338,10 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
     unsigned char* smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
+    __shared__ int drain_s;          // never raised: drain waits end on completion or on the time limit, not on an abort
     __shared__ int decision_s[2];
     volatile int* abort_flag = &abort_s;
+    volatile int* drain_flag = &drain_s;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t rank = blockIdx.x % p.CL;          // slice of 128 components within the group
@@ -349,6 +354,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
 
     if (tid == 0) {
         abort_s = 0;
+        drain_s = 0;
         decision_s[0] = 0;
         decision_s[1] = 0;
         bar_init(BAR(B_YFULL0), 1);    bar_init(BAR(B_YFULL1), 1);      // one arrive.expect_tx by the producer + the TMA bytes
@@ -655,7 +661,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                 // publish (m, s) of this CTA's 128 components, then collect the group's
                 const uint32_t tag = (uint32_t)(i + 1);
                 XSlot* ring = xg + (size_t)(i & 3) * p.CL * 64 + p0 + pt;
-                xslot_write(ring + rank * 64, mc, sc, tag);
+                // (test hook: one CTA stays silent for the first tile, so that its peers' bounded waits run out)
+                if (!(p.test_silent_rank == (int)rank && cluster_id == 0 && i == 0)) xslot_write(ring + rank * 64, mc, sc, tag);
                 TOC(tk_, 3);
                 float2 e[8];
 #ifdef FLASHGMM_DEBUG
@@ -819,7 +826,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
         // On an abort the consumer may never wait for the last loads: they must have landed before the CTA may exit.
         if (!ok || *abort_flag) {
             for (int64_t i = (issued > 2 ? issued - 2 : 0); i < issued; ++i) {
-                if (lane == 0) bar_wait(BAR(B_YFULL0 + (int)(i & 1)), (uint32_t)((i >> 1) & 1), abort_flag, p.status, false);
+                if (lane == 0) bar_wait(BAR(B_YFULL0 + (int)(i & 1)), (uint32_t)((i >> 1) & 1), drain_flag, p.status, false);
                 __syncwarp();
             }
         }
@@ -1006,7 +1013,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
         // drain: every MMA issued by this warp has completed before TMEM is released
         if (elect_one()) mma_commit(BAR(B_FINAL));
         __syncwarp();
-        wait_all(BAR(B_FINAL), 0);
+        if (lane == 0) bar_wait(BAR(B_FINAL), 0, drain_flag, p.status, false);      // also after an abort
+        __syncwarp();
+        fence_after();
     }
 
     // teardown: everybody meets, peers are done with this CTA's shared memory, TMEM is released
@@ -1256,6 +1265,13 @@ extern "C" void gmm_debug_set_clk(long long* p) { g_tc_clk = p; }
 #endif
 
 int g_tc_order = 2;
+// test hooks of the time-out path (see tc_set_test_hooks)
+int g_tc_test_silent_rank = -1;
+unsigned long long g_tc_wait_limit_ns = 2000000000ull, g_tc_wait_limit_set = 2000000000ull;
+void tc_set_test_hooks(int silent_rank, unsigned long long wait_limit_ns) {
+    g_tc_test_silent_rank = silent_rank;
+    g_tc_wait_limit_ns = wait_limit_ns ? wait_limit_ns : 2000000000ull;
+}
 void tc_set_order(int o) { g_tc_order = o; }
 
 bool tc_supports(int D, int K) { return D >= 1 && D <= 128 && K >= 1 && K <= 1024; }
@@ -1343,6 +1359,13 @@ cudaError_t launch_em_tc(cudaStream_t s, const float* X, int64_t n, int D, int K
     p.X = X; p.n = n; p.D = D; p.K = K; p.CL = pl.CL; p.Q = Q; p.n_ks = pl.n_ks;
     p.flush = (flush_tiles < 2) ? 2 : (flush_tiles & ~1);
     p.order = g_tc_order;
+    p.test_silent_rank = g_tc_test_silent_rank;
+    if (g_tc_wait_limit_ns != g_tc_wait_limit_set) {
+        const cudaError_t ew = cudaMemcpyToSymbolAsync(c_wait_limit_ns, &g_tc_wait_limit_ns, sizeof(unsigned long long), 0,
+                                                       cudaMemcpyHostToDevice, s);
+        if (ew != cudaSuccess) return ew;
+        g_tc_wait_limit_set = g_tc_wait_limit_ns;
+    }
     p.phi_img = tb.phi_img; p.plo_img = tb.plo_img; p.tk = tb.tk; p.ck = tb.ck;
     p.illb = tb.illb; p.flags = tb.flags; p.mu = mu; p.w2 = w2; p.c2 = c2;
     p.partial = tb.partial; p.llpart = tb.llpart; p.status = status;

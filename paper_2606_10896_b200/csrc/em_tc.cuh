@@ -39,6 +39,9 @@ struct TcBuffers {
 
 bool tc_supports(int D, int K);
 void tc_set_order(int o);   // MMA issue order: 0 = pairs E E M M, 1 = interleaved M(i) E(i+2), 2 = whichever of E(i+2), M(i+1) is ready first (default)
+// Time-out test: CTA `silent_rank` of group 0 never publishes its exchange slot for tile 0 (-1: off), and every device-side
+// wait gives up after wait_limit_ns (0: the default 2 s).  Process-wide, like tc_set_order.
+void tc_set_test_hooks(int silent_rank, unsigned long long wait_limit_ns);
 TcPlan tc_plan(int D, int K, int num_sms);
 size_t tc_scratch_bytes(int D, int K);
 cudaError_t tc_max_clusters(int D, int K, int* out);

@@ -369,6 +369,11 @@ int gmm_create(gmm_ctx** out, int device, void* cuda_stream) {
         const long long v = std::atoll(e);
         if (v >= 64 && v <= TC_YPOINTS) ctx->tc_piece = v / 64 * 64;
     }
+    {   // test hooks of the bounded-wait path, process-wide and set at every create like the issue order
+        const char* r = std::getenv("GMM_TC_TEST_SILENT_RANK");
+        const char* w = std::getenv("GMM_TC_TEST_WAIT_MS");
+        tc_set_test_hooks(r ? std::atoi(r) : -1, w ? (unsigned long long)std::atoll(w) * 1000000ull : 0ull);
+    }
     {   // the issue order is process-wide: every create sets it, so a context never inherits an earlier context's choice
         const char* e = std::getenv("GMM_TC_ORDER");
         tc_set_order(e ? std::atoi(e) : 2);

@@ -126,6 +126,32 @@ def test_tensor_path_accumulates_over_pieces(fg, monkeypatch):
         _teacher_forced(fg, c, synth.sample_host(spec), spec, 2, paths=[fg.GMM_PATH_TENSOR])
 
 
+def test_bounded_wait_runs_out_and_the_gpu_stays_usable(fg, monkeypatch):
+    # Every device-side wait of the tensor path is bounded.  A test hook makes one CTA of the first group keep its
+    # exchange slot of the first tile empty (a flag that nothing sets); with the limit shortened to 100 ms its peers'
+    # waits run out, every role of those CTAs leaves through the abort path, the kernel ends by itself and the call
+    # returns GMM_ETIMEOUT.  Nothing faults or hangs: a fresh context then computes the same step correctly.
+    spec = synth.CONFIGS[2].with_n(3000)
+    X = synth.sample_host(spec)
+    pi0, mu0, var0 = synth.init_params(X, spec)
+    p32, m32, v32 = pi0.astype(np.float32), mu0.astype(np.float32), var0.astype(np.float32)
+    monkeypatch.setenv("GMM_TC_TEST_SILENT_RANK", "3")
+    monkeypatch.setenv("GMM_TC_TEST_WAIT_MS", "100")
+    with fg.Context(0) as c:
+        c.gmm_set_path(fg.GMM_PATH_TENSOR)
+        with pytest.raises(fg.GmmError) as err:
+            _gpu_step(c, _t(X), p32, m32, v32)
+        assert err.value.code == fg.GMM_ETIMEOUT
+    monkeypatch.delenv("GMM_TC_TEST_SILENT_RANK")
+    monkeypatch.delenv("GMM_TC_TEST_WAIT_MS")
+    ref = orc.em_step(X, p32, m32, v32)
+    with fg.Context(0) as c:
+        c.gmm_set_path(fg.GMM_PATH_TENSOR)
+        got = _gpu_step(c, _t(X), p32, m32, v32)
+        assert abs(got[3] - ref[3]) <= 1e-5 * abs(ref[3])
+        assert_stats_close(len(X), data_scale(X), got[:3], ref[:3], "after a timed-out call")
+
+
 def test_config2_free_running_30_iterations(fg, ctx):
     """Config 2 as specified (N = 100,000, D = 128, K = 1024, 30 iterations): both sides iterate freely from the same
     initial parameters; the log-likelihood traces agree to 1e-4 relative at every iteration."""

@@ -131,6 +131,22 @@ int gmm_assign_topm(gmm_ctx* ctx, const float* X, int64_t N, int D, int K,
                     const float* pi, const float* mu, const float* var, int m,
                     int32_t* idx, float* resp);
 
+/* IVF posting lists from the top-m assignment (paper Section 4.2: every vector is stored with the cluster of its highest
+ * responsibility; Section 4.3, multi-assignment: with at most two clusters, the top clusters whose responsibility
+ * exceeds tau = 1/K).  The rule implemented: choice 0 of a vector is always taken; choices 1 .. max_lists-1 are taken
+ * in order while resp > tau (strictly); a negative index ends a vector's list.
+ *   idx [N x m] int32, resp [N x m] float32: device, as written by gmm_assign_topm (descending responsibility).
+ *   tau: threshold; <= 0 selects the paper's 1/K.   max_lists: 1 (hard assignment) .. m (the paper uses 2).
+ *   offsets [K + 1] int64, device out: list k holds items[offsets[k] .. offsets[k+1]).
+ *   items  int32, device out, capacity >= N * max_lists entries: vector indices, ascending inside every list.
+ *   total (host out, may be NULL): offsets[K];  mean_lists (host out, may be NULL): total / N, the paper's average
+ *   number of posting lists per vector (Section 5, multi-assignment analysis).
+ * Deterministic (no atomics on the output); scratch O(K), independent of N.  Limits: N < 2^31, K <= 8192 (otherwise
+ * GMM_EUNSUPPORTED).  Synchronises the stream. */
+int gmm_build_posting_lists(gmm_ctx* ctx, const int32_t* idx, const float* resp, int64_t N, int m, int K,
+                            float tau, int max_lists, int64_t* offsets, int32_t* items,
+                            int64_t* total, double* mean_lists);
+
 /* The statistics of gmm_em_step for callers that cannot allocate device memory.  (The paper has no counterpart of
  * this entry point; it exists for the library's users.)
  *

@@ -85,6 +85,8 @@ struct gmm_ctx {
     unsigned char* scratch = nullptr;
     size_t scratch_bytes = 0;
     int capD = 0, capK = 0;
+    void* pl_scratch = nullptr;      // posting-list builder: counters per (range of vectors, cluster)
+    size_t pl_scratch_bytes = 0;
     bool capPlanes = false;    // the scratch layout in force includes the tensor path's planes of Y
     ScratchLayout lay{};
     int tc_Q = 0;              // resident clusters of the tensor-path kernel for (capD, capK)
@@ -393,6 +395,7 @@ int gmm_destroy(gmm_ctx* ctx) {
         if (ctx->ev_done[b]) cudaEventDestroy(ctx->ev_done[b]);
     }
     if (ctx->hparams) cudaFree(ctx->hparams);
+    if (ctx->pl_scratch) cudaFree(ctx->pl_scratch);
     if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
     if (ctx->ev_created)
         for (int i = 0; i < EVENT_POOL; ++i) {
@@ -652,6 +655,42 @@ int gmm_reset_counters(gmm_ctx* ctx) {
     ctx->prof_ms = 0.0;
     ctx->prof_launches = 0;
     ctx->ev_used = 0;
+    return GMM_OK;
+}
+
+int gmm_build_posting_lists(gmm_ctx* ctx, const int32_t* idx, const float* resp, int64_t N, int m, int K, float tau,
+                            int max_lists, int64_t* offsets, int32_t* items, int64_t* total, double* mean_lists) {
+    if (!ctx) return GMM_EINVAL;
+    DeviceGuard g(ctx->device);
+    if (!idx || !resp || !offsets || !items) return fail(ctx, GMM_EINVAL, "null pointer argument");
+    if (N < 1 || K < 1) return fail(ctx, GMM_EINVAL, "N and K must be >= 1 (got N=%lld K=%d)", (long long)N, K);
+    if (m < 1 || m > GMM_MAX_TOPM) return fail(ctx, GMM_EINVAL, "m must be in [1, %d] (got %d)", GMM_MAX_TOPM, m);
+    if (max_lists < 1 || max_lists > m) return fail(ctx, GMM_EINVAL, "max_lists must be in [1, m] (got %d, m=%d)", max_lists, m);
+    if (N >= ((int64_t)1 << 31)) return fail(ctx, GMM_EUNSUPPORTED, "N must be below 2^31 (vector indices are int32)");
+    if (K > PL_MAX_K) return fail(ctx, GMM_EUNSUPPORTED, "K must be <= %d for the posting-list builder (got %d)", PL_MAX_K, K);
+    if (!(tau > 0.f)) tau = 1.0f / (float)K;                 // also for NaN
+    const size_t need = pl_scratch_bytes(K);
+    if (need > ctx->pl_scratch_bytes) {
+        if (ctx->pl_scratch) {
+            CU(cudaStreamSynchronize(ctx->stream));
+            CU(cudaFree(ctx->pl_scratch));
+            ctx->pl_scratch = nullptr;
+            ctx->pl_scratch_bytes = 0;
+        }
+        cudaError_t e = cudaMalloc(&ctx->pl_scratch, need);
+        if (e != cudaSuccess) {
+            cudaGetLastError();
+            return fail(ctx, GMM_ENOMEM, "cannot allocate %zu bytes for the posting-list counters: %s", need, cudaGetErrorString(e));
+        }
+        ctx->pl_scratch_bytes = need;
+    }
+    KL(launch_posting_lists(ctx->stream, idx, resp, N, m, K, tau, max_lists, ctx->pl_scratch, offsets, items));
+    ctx->launches += 4;        // launch_posting_lists enqueues five kernels
+    int64_t tot = 0;
+    CU(cudaMemcpyAsync(&tot, offsets + K, sizeof(int64_t), cudaMemcpyDeviceToHost, ctx->stream));
+    CU(cudaStreamSynchronize(ctx->stream));
+    if (total) *total = tot;
+    if (mean_lists) *mean_lists = (double)tot / (double)N;
     return GMM_OK;
 }
 

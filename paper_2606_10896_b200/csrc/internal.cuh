@@ -52,4 +52,12 @@ cudaError_t launch_finalize(cudaStream_t s, int64_t N, int D, int K, const doubl
 cudaError_t launch_finalize_isotropic(cudaStream_t s, int64_t N, int D, int K, const double* Nk, const double* S1,
                                       const double* S2, float var_floor, float* pi, float* mu, float* var);
 
+// ---- IVF posting lists from the top-m assignment (paper Sections 4.2-4.3) ---------------------------------------
+constexpr int PL_MAX_BLOCKS = 1024;       // the vectors are cut into at most this many contiguous ranges
+constexpr int PL_MAX_K = 8192;            // one 32-bit cursor per cluster in shared memory
+size_t pl_scratch_bytes(int K);
+// offsets[K + 1] (device), items[>= n * max_lists] (device); scratch of pl_scratch_bytes(K) bytes
+cudaError_t launch_posting_lists(cudaStream_t s, const int32_t* idx, const float* resp, int64_t n, int m, int K, float tau,
+                                 int max_lists, void* scratch, int64_t* offsets, int32_t* items);
+
 }  // namespace fg

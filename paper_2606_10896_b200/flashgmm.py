@@ -51,6 +51,9 @@ EXPORTS = {
     "gmm_assign_topm": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_int,
                                        ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int,
                                        ctypes.c_void_p, ctypes.c_void_p]),
+    "gmm_build_posting_lists": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int,
+                                               ctypes.c_int, ctypes.c_float, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p,
+                                               ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_double)]),
     "gmm_em_step_static": (ctypes.c_int, [ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int,
                                           ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                           ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
@@ -281,3 +284,20 @@ class Context:
                                  _dev(idx, torch.int32, (N, m), "idx"), _dev(resp, torch.float32, (N, m), "resp"))
         self._check(rc)
         return idx, resp
+
+    def gmm_build_posting_lists(self, idx, resp, K, tau=None, max_lists=2, out=None):
+        """Posting lists from a top-m assignment: (offsets int64 [K + 1], items int32 [N * max_lists], total, mean lists
+        per vector); list k is items[offsets[k]:offsets[k + 1]], ascending.  tau None selects 1 / K."""
+        N, m = idx.shape
+        if out is None:
+            offsets = torch.empty(int(K) + 1 if K >= 0 else 1, dtype=torch.int64, device=idx.device)
+            items = torch.empty(max(1, N * max(1, int(max_lists))), dtype=torch.int32, device=idx.device)
+        else:
+            offsets, items = out
+        total, mean = ctypes.c_int64(0), ctypes.c_double(0.0)
+        rc = lib.gmm_build_posting_lists(self._h, _dev(idx, torch.int32, (N, m), "idx"), _dev(resp, torch.float32, (N, m), "resp"),
+                                         N, m, int(K), float(tau) if tau is not None else 0.0, int(max_lists),
+                                         ctypes.c_void_p(offsets.data_ptr()), ctypes.c_void_p(items.data_ptr()),
+                                         ctypes.byref(total), ctypes.byref(mean))
+        self._check(rc)
+        return offsets, items, int(total.value), float(mean.value)

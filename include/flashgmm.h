@@ -147,6 +147,20 @@ int gmm_build_posting_lists(gmm_ctx* ctx, const int32_t* idx, const float* resp,
                             float tau, int max_lists, int64_t* offsets, int32_t* items,
                             int64_t* total, double* mean_lists);
 
+/* One Lloyd (k-means) iteration, the warm start the paper runs before its EM iterations (Section 5, experimental setup:
+ * 10 iterations of k-means, then Flash-GMM).  Assignment: every point goes to the centroid at the smallest squared
+ * Euclidean distance (direct differences in fp32; ties to the smaller index).  Update: a centroid becomes the mean of its
+ * points (float64 sums in a fixed order); a centroid without points keeps its position.
+ *   X [N x D], centroids [K x D]: device, row-major fp32.
+ *   assign [N] int32, device out: the index of each point's nearest centroid.
+ *   work [2 N] int32, device scratch owned by the caller (the library holds no O(N) memory).
+ *   centroids_out [K x D] fp32, device out (may be the same array as centroids).
+ *   counts [K] int64, device out, may be NULL: points per centroid.
+ *   inertia (host out, may be NULL): sum over the points of the squared distance to their (input) centroid.
+ * Deterministic (no atomics).  Limits: N < 2^31, K <= 8192 (otherwise GMM_EUNSUPPORTED).  Synchronises the stream. */
+int gmm_kmeans_step(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const float* centroids,
+                    int32_t* assign, int32_t* work, float* centroids_out, int64_t* counts, double* inertia);
+
 /* The statistics of gmm_em_step for callers that cannot allocate device memory.  (The paper has no counterpart of
  * this entry point; it exists for the library's users.)
  *

@@ -86,6 +86,8 @@ struct gmm_ctx {
     size_t scratch_bytes = 0;
     int capD = 0, capK = 0;
     void* pl_scratch = nullptr;      // posting-list builder: counters per (range of vectors, cluster)
+    void* km_scratch = nullptr;      // k-means step: list offsets, per-segment float64 sums
+    size_t km_scratch_bytes = 0;
     size_t pl_scratch_bytes = 0;
     bool capPlanes = false;    // the scratch layout in force includes the tensor path's planes of Y
     ScratchLayout lay{};
@@ -396,6 +398,7 @@ int gmm_destroy(gmm_ctx* ctx) {
     }
     if (ctx->hparams) cudaFree(ctx->hparams);
     if (ctx->pl_scratch) cudaFree(ctx->pl_scratch);
+    if (ctx->km_scratch) cudaFree(ctx->km_scratch);
     if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
     if (ctx->ev_created)
         for (int i = 0; i < EVENT_POOL; ++i) {
@@ -658,6 +661,26 @@ int gmm_reset_counters(gmm_ctx* ctx) {
     return GMM_OK;
 }
 
+namespace {
+// grows *buf to at least `need` bytes (contents are not kept)
+int grow_buffer(gmm_ctx* ctx, void** buf, size_t* have, size_t need, const char* what) {
+    if (need <= *have) return GMM_OK;
+    if (*buf) {
+        CU(cudaStreamSynchronize(ctx->stream));
+        CU(cudaFree(*buf));
+        *buf = nullptr;
+        *have = 0;
+    }
+    cudaError_t e = cudaMalloc(buf, need);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return fail(ctx, GMM_ENOMEM, "cannot allocate %zu bytes for %s: %s", need, what, cudaGetErrorString(e));
+    }
+    *have = need;
+    return GMM_OK;
+}
+}  // namespace
+
 int gmm_build_posting_lists(gmm_ctx* ctx, const int32_t* idx, const float* resp, int64_t N, int m, int K, float tau,
                             int max_lists, int64_t* offsets, int32_t* items, int64_t* total, double* mean_lists) {
     if (!ctx) return GMM_EINVAL;
@@ -669,21 +692,7 @@ int gmm_build_posting_lists(gmm_ctx* ctx, const int32_t* idx, const float* resp,
     if (N >= ((int64_t)1 << 31)) return fail(ctx, GMM_EUNSUPPORTED, "N must be below 2^31 (vector indices are int32)");
     if (K > PL_MAX_K) return fail(ctx, GMM_EUNSUPPORTED, "K must be <= %d for the posting-list builder (got %d)", PL_MAX_K, K);
     if (!(tau > 0.f)) tau = 1.0f / (float)K;                 // also for NaN
-    const size_t need = pl_scratch_bytes(K);
-    if (need > ctx->pl_scratch_bytes) {
-        if (ctx->pl_scratch) {
-            CU(cudaStreamSynchronize(ctx->stream));
-            CU(cudaFree(ctx->pl_scratch));
-            ctx->pl_scratch = nullptr;
-            ctx->pl_scratch_bytes = 0;
-        }
-        cudaError_t e = cudaMalloc(&ctx->pl_scratch, need);
-        if (e != cudaSuccess) {
-            cudaGetLastError();
-            return fail(ctx, GMM_ENOMEM, "cannot allocate %zu bytes for the posting-list counters: %s", need, cudaGetErrorString(e));
-        }
-        ctx->pl_scratch_bytes = need;
-    }
+    CHECK(grow_buffer(ctx, &ctx->pl_scratch, &ctx->pl_scratch_bytes, pl_scratch_bytes(K), "the posting-list counters"));
     KL(launch_posting_lists(ctx->stream, idx, resp, N, m, K, tau, max_lists, ctx->pl_scratch, offsets, items));
     ctx->launches += 4;        // launch_posting_lists enqueues five kernels
     int64_t tot = 0;
@@ -691,6 +700,43 @@ int gmm_build_posting_lists(gmm_ctx* ctx, const int32_t* idx, const float* resp,
     CU(cudaStreamSynchronize(ctx->stream));
     if (total) *total = tot;
     if (mean_lists) *mean_lists = (double)tot / (double)N;
+    return GMM_OK;
+}
+
+int gmm_kmeans_step(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const float* centroids, int32_t* assign,
+                    int32_t* work, float* centroids_out, int64_t* counts, double* inertia) {
+    CHECK(check_shape(ctx, N, D, K));
+    CHECK(check_ptr(ctx, X, 4, "X"));
+    CHECK(check_ptr(ctx, centroids, 4, "centroids"));
+    CHECK(check_ptr(ctx, assign, 4, "assign"));
+    CHECK(check_ptr(ctx, work, 4, "work"));
+    CHECK(check_ptr(ctx, centroids_out, 4, "centroids_out"));
+    if (N >= ((int64_t)1 << 31)) return fail(ctx, GMM_EUNSUPPORTED, "N must be below 2^31 (point indices are int32)");
+    if (K > PL_MAX_K) return fail(ctx, GMM_EUNSUPPORTED, "K must be <= %d for the k-means step (got %d)", PL_MAX_K, K);
+    DeviceGuard g(ctx->device);
+    CHECK(ensure_scratch(ctx, D, K));
+    CHECK(grow_buffer(ctx, &ctx->pl_scratch, &ctx->pl_scratch_bytes, pl_scratch_bytes(K), "the posting-list counters"));
+    CHECK(grow_buffer(ctx, &ctx->km_scratch, &ctx->km_scratch_bytes, km_scratch_bytes(D, K), "the k-means partial sums"));
+    // nearest centroid = top-1 component of a unit-variance, equal-weight mixture
+    KL(launch_kmeans_unit_params(ctx->stream, D, K, ctx->w2(), ctx->c2d()));
+    float* resp = reinterpret_cast<float*>(work);                 // [N], not used afterwards except as the builder's input
+    int32_t* items = work + N;                                    // [N]
+    for (int64_t off = 0; off < N; off += SUPER_TILE) {
+        const int64_t cnt = (N - off < SUPER_TILE) ? (N - off) : SUPER_TILE;
+        KL(launch_topm_fp32(ctx->stream, X + off * D, cnt, D, K, centroids, ctx->w2(), ctx->c2d(), 1, assign + off, resp + off));
+    }
+    // the points of every cluster in ascending order, then fixed-order float64 sums
+    KL(launch_posting_lists(ctx->stream, assign, resp, N, 1, K, 1.0f, 1, ctx->pl_scratch, km_offsets(ctx->km_scratch), items));
+    KL(launch_kmeans_update(ctx->stream, X, D, K, centroids, items, ctx->km_scratch, centroids_out, counts));
+    ctx->launches += 5;
+    const int slot = 0;
+    CU(cudaMemsetAsync(&ctx->result()->ll[slot], 0, 8, ctx->stream));
+    KL(launch_reduce_ll(ctx->stream, km_inertia_k(ctx->km_scratch, D, K), K, &ctx->result()->ll[slot], false));
+    double v = 0.0;
+    CU(cudaMemcpyAsync(&v, &ctx->result()->ll[slot], sizeof(double), cudaMemcpyDeviceToHost, ctx->stream));
+    CU(cudaStreamSynchronize(ctx->stream));
+    if (inertia) *inertia = v;
+    ctx->last_path = GMM_PATH_FP32;
     return GMM_OK;
 }
 

@@ -60,4 +60,12 @@ size_t pl_scratch_bytes(int K);
 cudaError_t launch_posting_lists(cudaStream_t s, const int32_t* idx, const float* resp, int64_t n, int m, int K, float tau,
                                  int max_lists, void* scratch, int64_t* offsets, int32_t* items);
 
+// ---- one Lloyd (k-means) iteration: the paper's warm start (Section 5) -----------------------------------------------
+size_t km_scratch_bytes(int D, int K);
+int64_t* km_offsets(void* scratch);                     // [K + 1] inside the scratch: the posting-list offsets go here
+double* km_inertia_k(void* scratch, int D, int K);      // [K] per-cluster inertia, written by launch_kmeans_update
+cudaError_t launch_kmeans_unit_params(cudaStream_t s, int D, int K, float* w2, double* c2d);
+cudaError_t launch_kmeans_update(cudaStream_t s, const float* X, int D, int K, const float* cent_in, const int32_t* items,
+                                 void* scratch, float* cent_out, int64_t* counts);
+
 }  // namespace fg

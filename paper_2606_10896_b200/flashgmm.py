@@ -54,6 +54,9 @@ EXPORTS = {
     "gmm_build_posting_lists": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int,
                                                ctypes.c_int, ctypes.c_float, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p,
                                                ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_double)]),
+    "gmm_kmeans_step": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_int, ctypes.c_void_p,
+                                       ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                       ctypes.POINTER(ctypes.c_double)]),
     "gmm_em_step_static": (ctypes.c_int, [ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int,
                                           ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                           ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
@@ -301,3 +304,23 @@ class Context:
                                          ctypes.byref(total), ctypes.byref(mean))
         self._check(rc)
         return offsets, items, int(total.value), float(mean.value)
+
+    def gmm_kmeans_step(self, X, centroids, out=None, work=None):
+        """One Lloyd iteration: (assign int32 [N], new centroids float32 [K, D], counts int64 [K], inertia)."""
+        N, D = X.shape
+        K = centroids.shape[0]
+        if out is None:
+            assign = torch.empty(N, dtype=torch.int32, device=X.device)
+            new = torch.empty((K, D), dtype=torch.float32, device=X.device)
+            counts = torch.empty(K, dtype=torch.int64, device=X.device)
+        else:
+            assign, new, counts = out
+        if work is None:
+            work = torch.empty(2 * N, dtype=torch.int32, device=X.device)
+        inertia = ctypes.c_double(0.0)
+        rc = lib.gmm_kmeans_step(self._h, _dev(X, torch.float32, (N, D), "X"), N, D, K,
+                                 _dev(centroids, torch.float32, (K, D), "centroids"), _dev(assign, torch.int32, (N,), "assign"),
+                                 _dev(work, torch.int32, (2 * N,), "work"), _dev(new, torch.float32, (K, D), "centroids_out"),
+                                 ctypes.c_void_p(counts.data_ptr()), ctypes.byref(inertia))
+        self._check(rc)
+        return assign, new, counts, float(inertia.value)

@@ -1047,48 +1047,65 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
 // [16 ks + 8, 16 ks + 16) = (s x)^2 + kap, i.e. the column order of the E-step contraction.  One thread converts one
 // (point, k-step) unit and writes 32 contiguous bytes per plane; 16 consecutive threads write one 512-byte row.
 // Rows n .. rows_padded - 1 are written as zeros so that the last tile's loads need no out-of-bounds handling.
+__device__ __forceinline__ void tc_load_unit(const float* __restrict__ X, int64_t n, int D, bool vec_ok, int64_t u, int64_t units,
+                                             float (&x)[8]) {
+    const int64_t row = u >> 4;
+    const int d0 = (int)(u & 15) * 8;
+    if (u < units && row < n && vec_ok && d0 + 8 <= D) {
+        const float4 a = __ldg(reinterpret_cast<const float4*>(X + row * D + d0));
+        const float4 b = __ldg(reinterpret_cast<const float4*>(X + row * D + d0 + 4));
+        x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
+    } else {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) x[j] = (u < units && row < n && d0 + j < D) ? __ldg(X + row * D + d0 + j) : 0.f;
+    }
+}
+
+__device__ __forceinline__ void tc_store_unit(const float (&x)[8], int64_t n, const float* __restrict__ sd,
+                                              const float* __restrict__ kap, int64_t u, unsigned char* __restrict__ yhi,
+                                              unsigned char* __restrict__ ylo) {
+    const int64_t row = u >> 4;
+    const int ks = (int)(u & 15), d0 = ks * 8;
+    uint32_t xh[4], xl[4], qh[4], ql[4];
+#pragma unroll
+    for (int j = 0; j < 8; j += 2) {
+        float u0 = x[j] * __ldg(sd + d0 + j), u1 = x[j + 1] * __ldg(sd + d0 + j + 1);
+        u0 = fminf(fmaxf(u0, -240.f), 240.f);
+        u1 = fminf(fmaxf(u1, -240.f), 240.f);
+        float q0 = fmaf(u0, u0, __ldg(kap + d0 + j)), q1 = fmaf(u1, u1, __ldg(kap + d0 + j + 1));
+        if (row >= n) { q0 = 0.f; q1 = 0.f; }
+        const __half2 h = __floats2half2_rn(u0, u1);
+        const float2 hf = __half22float2(h);
+        const __half2 g2 = __floats2half2_rn(u0 - hf.x, u1 - hf.y);
+        const __half2 sq = __floats2half2_rn(q0, q1);
+        const float2 sf = __half22float2(sq);
+        const __half2 t2 = __floats2half2_rn(q0 - sf.x, q1 - sf.y);
+        xh[j / 2] = *reinterpret_cast<const uint32_t*>(&h);
+        xl[j / 2] = *reinterpret_cast<const uint32_t*>(&g2);
+        qh[j / 2] = *reinterpret_cast<const uint32_t*>(&sq);
+        ql[j / 2] = *reinterpret_cast<const uint32_t*>(&t2);
+    }
+    uint4* oh = reinterpret_cast<uint4*>(yhi + row * 512 + ks * 32);
+    uint4* ol = reinterpret_cast<uint4*>(ylo + row * 512 + ks * 32);
+    oh[0] = make_uint4(xh[0], xh[1], xh[2], xh[3]);
+    oh[1] = make_uint4(qh[0], qh[1], qh[2], qh[3]);
+    ol[0] = make_uint4(xl[0], xl[1], xl[2], xl[3]);
+    ol[1] = make_uint4(ql[0], ql[1], ql[2], ql[3]);
+}
+
 __global__ void __launch_bounds__(256) tc_transform_kernel(const float* __restrict__ X, int64_t n, int64_t rows_padded, int D,
                                                            const float* __restrict__ sd, const float* __restrict__ kap,
                                                            unsigned char* __restrict__ yhi, unsigned char* __restrict__ ylo) {
     const bool vec_ok = (D % 4 == 0) && ((reinterpret_cast<uintptr_t>(X) & 15) == 0);
     const int64_t units = rows_padded * 16;
-    for (int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; u < units; u += (int64_t)gridDim.x * blockDim.x) {
-        const int64_t row = u >> 4;
-        const int ks = (int)(u & 15), d0 = ks * 8;
-        float x[8];
-        if (row < n && vec_ok && d0 + 8 <= D) {
-            const float4 a = __ldg(reinterpret_cast<const float4*>(X + row * D + d0));
-            const float4 b = __ldg(reinterpret_cast<const float4*>(X + row * D + d0 + 4));
-            x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
-        } else {
-#pragma unroll
-            for (int j = 0; j < 8; ++j) x[j] = (row < n && d0 + j < D) ? __ldg(X + row * D + d0 + j) : 0.f;
-        }
-        uint32_t xh[4], xl[4], qh[4], ql[4];
-#pragma unroll
-        for (int j = 0; j < 8; j += 2) {
-            float u0 = x[j] * __ldg(sd + d0 + j), u1 = x[j + 1] * __ldg(sd + d0 + j + 1);
-            u0 = fminf(fmaxf(u0, -240.f), 240.f);
-            u1 = fminf(fmaxf(u1, -240.f), 240.f);
-            float q0 = fmaf(u0, u0, __ldg(kap + d0 + j)), q1 = fmaf(u1, u1, __ldg(kap + d0 + j + 1));
-            if (row >= n) { q0 = 0.f; q1 = 0.f; }
-            const __half2 h = __floats2half2_rn(u0, u1);
-            const float2 hf = __half22float2(h);
-            const __half2 g2 = __floats2half2_rn(u0 - hf.x, u1 - hf.y);
-            const __half2 sq = __floats2half2_rn(q0, q1);
-            const float2 sf = __half22float2(sq);
-            const __half2 t2 = __floats2half2_rn(q0 - sf.x, q1 - sf.y);
-            xh[j / 2] = *reinterpret_cast<const uint32_t*>(&h);
-            xl[j / 2] = *reinterpret_cast<const uint32_t*>(&g2);
-            qh[j / 2] = *reinterpret_cast<const uint32_t*>(&sq);
-            ql[j / 2] = *reinterpret_cast<const uint32_t*>(&t2);
-        }
-        uint4* oh = reinterpret_cast<uint4*>(yhi + row * 512 + ks * 32);
-        uint4* ol = reinterpret_cast<uint4*>(ylo + row * 512 + ks * 32);
-        oh[0] = make_uint4(xh[0], xh[1], xh[2], xh[3]);
-        oh[1] = make_uint4(qh[0], qh[1], qh[2], qh[3]);
-        ol[0] = make_uint4(xl[0], xl[1], xl[2], xl[3]);
-        ol[1] = make_uint4(ql[0], ql[1], ql[2], ql[3]);
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    // two units per step, both loads issued before the first store: twice the bytes in flight per thread
+    for (int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; u < units; u += 2 * stride) {
+        float xa[8], xb[8];
+        tc_load_unit(X, n, D, vec_ok, u, units, xa);
+        tc_load_unit(X, n, D, vec_ok, u + stride, units, xb);
+        tc_store_unit(xa, n, sd, kap, u, yhi, ylo);
+        if (u + stride < units) tc_store_unit(xb, n, sd, kap, u + stride, yhi, ylo);
     }
 }
 

@@ -1,0 +1,547 @@
+// Top-m assignment on the tensor cores (sm_100a, tcgen05 + TMEM): paper Sections 4.2-4.3 (hard assignment and
+// multi-assignment read the largest responsibilities of every vector), computed from the same expanded quadratic form
+// as the E-step of Algorithm 1.
+//
+// Two kernels per piece of at most TC_YPOINTS points, after tc_transform_kernel has written the fp16 planes of Y:
+//
+//   assign_tc_kernel   lanes of TMEM = POINTS (the E+M tile kernel has lanes = components because its M-step needs that;
+//                      selection wants the opposite: one thread owns one point and walks over the components, so neither
+//                      the log-sum-exp nor the selection needs a single cross-lane operation or an exchange between CTAs).
+//                      A persistent CTA takes tiles of 128 points: the tile's two planes of Y stay in shared memory (A operand,
+//                      128 KB) while the coefficient planes P_hi, P_lo of all K components stream through a ring of
+//                      32 KB stages (B operand: 128 components x 64 columns x 2 planes, from L2 by TMA).  Per chunk of 128
+//                      components: logits (approximate, 22-bit operands) = Y_hi P_lo + Y_lo P_hi + Y_hi P_hi in a 128-column TMEM
+//                      buffer; two such buffers, one per softmax warpgroup, alternate.  A softmax thread keeps for its point
+//                      the running (max, sum) of the log-sum-exp and the LIST largest logits with their indices, and
+//                      writes one record per tile.
+//   assign_refine_kernel  one warp per point: merges the records of the two warpgroups, recomputes the LIST - 1 best
+//                      candidates EXACTLY (fp32 direct differences, the arithmetic of the FP32 path), corrects the
+//                      log-sum-exp by the difference between exact and approximate candidate terms, orders by the exact
+//                      values (ties to the smaller index) and writes the top m.  The selection is certain when the m-th
+//                      exact value clears the best non-candidate's approximate value by more than the error bound of the
+//                      approximation; otherwise (near ties, exact ties, fewer than m finite candidates) the warp
+//                      walks over all K components exactly.
+#include "internal.cuh"
+#include "em_tc.cuh"
+
+#define TC_WAIT_LIMIT_NS 2000000000ull
+#include "tc_prims.cuh"
+
+namespace fg {
+
+namespace {
+
+constexpr int AT_POINTS = 128;               // points per tile = TMEM lanes
+constexpr int AT_COMPS = 128;                // components per chunk = MMA N
+constexpr int AT_THREADS = 320;              // 8 softmax warps, producer warp, MMA warp
+constexpr int AT_PRODUCER = 8, AT_MMA = 9;
+constexpr int AT_STAGES = 3;
+constexpr int AT_ATOM = 16384;               // 128 rows x 128 bytes
+constexpr int ASM_A = 0;                     // [plane][atom]: 2 x 4 x 16384
+constexpr int ASM_ALO = 4 * AT_ATOM;
+constexpr int ASM_B = 8 * AT_ATOM;           // stages x [plane]: 3 x 2 x 16384
+constexpr int ASM_BAR = ASM_B + AT_STAGES * 2 * AT_ATOM;
+constexpr int ASM_BYTES = ASM_BAR + 256 + 1024;      // barriers, alignment slack
+
+enum { AB_AFULL = 0, AB_AEMPTY = 4, AB_BFULL = 8, AB_BEMPTY = 8 + AT_STAGES, AB_LFULL = 8 + 2 * AT_STAGES,
+       AB_LEMPTY = AB_LFULL + 2, AB_FINAL = AB_LEMPTY + 2, AB_COUNT };
+
+struct AssignParams {
+    int64_t n;                 // points of this piece
+    int n_chunks, n_ks;
+    const float2* tkck;        // [n_chunks * 128] (t_k, c_k): log2 z = t_k * contraction + c_k
+    float* rec;                // [n][2][RECW] records (see assign_recw)
+    int* status;
+    const int* gate;           // the launch does nothing when gate[0] != 0 (too many ill-conditioned components: the FP32 kernels run instead)
+};
+
+constexpr int assign_recw(int LIST) { return (2 + 2 * LIST + 3) & ~3; }      // words per record: m, s, LIST values, LIST indices
+
+template <int LIST>
+__global__ void __launch_bounds__(AT_THREADS, 1)
+assign_tc_kernel(const AssignParams p, const __grid_constant__ CUtensorMap tm_yhi, const __grid_constant__ CUtensorMap tm_ylo,
+                 const __grid_constant__ CUtensorMap tm_phi, const __grid_constant__ CUtensorMap tm_plo) {
+    extern __shared__ unsigned char smem_raw[];
+    if (p.gate[0] != 0) return;                                     // uniform over the grid, before anything is allocated
+    unsigned char* smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int abort_s, drain_s;
+    volatile int* abort_flag = &abort_s;
+    volatile int* drain_flag = &drain_s;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int64_t ntiles = (p.n + AT_POINTS - 1) / AT_POINTS;
+    const int64_t ntl = ((int64_t)blockIdx.x < ntiles) ? (ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+    const int NC = p.n_chunks;
+    const int n_atoms = (p.n_ks + 3) >> 2;
+
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + ASM_BAR);
+    auto BAR = [&](int i) { return smem_u32(&bars[i]); };
+
+    if (tid == 0) {
+        abort_s = 0;
+        drain_s = 0;
+        for (int a = 0; a < 4; ++a) { bar_init(BAR(AB_AFULL + a), 1); bar_init(BAR(AB_AEMPTY + a), 1); }
+        for (int s = 0; s < AT_STAGES; ++s) { bar_init(BAR(AB_BFULL + s), 1); bar_init(BAR(AB_BEMPTY + s), 1); }
+        for (int b = 0; b < 2; ++b) { bar_init(BAR(AB_LFULL + b), 1); bar_init(BAR(AB_LEMPTY + b), 128); }
+        bar_init(BAR(AB_FINAL), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == AT_MMA) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(256) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    fence_before();
+    __syncthreads();
+    fence_after();
+    const uint32_t tmem = tmem_base_s;
+
+    if (warp < 8) {
+        // =========================== softmax / selection warps ===========================
+        // Warpgroup g takes the chunks c with c mod 2 = g (logits buffer g).  Thread = TMEM lane = point.
+        const int grp = warp >> 2, wq = warp & 3;
+        const uint32_t lane_addr = ((uint32_t)(wq * 32)) << 16;
+        const uint32_t tbuf = tmem + grp * AT_COMPS + lane_addr;
+        constexpr int RECW = assign_recw(LIST);
+        uint32_t uses = 0;                       // completed uses of this group's buffer
+        bool alive = true;
+        for (int64_t i = 0; i < ntl && alive; ++i) {
+            const int64_t row = (blockIdx.x + i * gridDim.x) * AT_POINTS + wq * 32 + lane;
+            float m_run = -1e30f, s_run = 0.f;          // finite start: a first block of -inf logits must not make NaN
+            float tv[LIST];
+            int ti[LIST];
+#pragma unroll
+            for (int j = 0; j < LIST; ++j) { tv[j] = -CUDART_INF_F; ti[j] = -1; }
+            for (int c = grp; c < NC; c += 2) {
+                // every lane waits itself, and the warp leaves together: the TMEM loads below are warp-wide instructions
+                const bool got = bar_wait(BAR(AB_LFULL + grp), uses & 1u, abort_flag, p.status, false);
+                if (!__all_sync(0xffffffffu, got)) { alive = false; break; }
+                fence_after();
+                ++uses;
+#pragma unroll 1
+                for (int sub = 0; sub < 4; ++sub) {
+                    uint32_t v[32];
+                    tmem_ld32(tbuf + sub * 32, v);
+                    tmem_wait_ld();
+                    if (sub == 3) {                     // the buffer's last columns are in registers: hand it back
+                        fence_before();
+                        bar_arrive(BAR(AB_LEMPTY + grp));
+                    }
+                    const int col0 = c * AT_COMPS + sub * 32;
+                    const float4* tc4 = reinterpret_cast<const float4*>(p.tkck + col0);
+                    float l[32];
+                    float bmax = -CUDART_INF_F;
+#pragma unroll
+                    for (int j = 0; j < 32; j += 2) {
+                        const float4 q = __ldg(tc4 + (j >> 1));          // (t, c) of two components; same address in every lane
+                        l[j] = fmaf(__uint_as_float(v[j]), q.x, q.y);
+                        l[j + 1] = fmaf(__uint_as_float(v[j + 1]), q.z, q.w);
+                        bmax = fmaxf(bmax, fmaxf(l[j], l[j + 1]));
+                    }
+                    if (bmax > m_run) {
+                        s_run *= fast_ex2(m_run - bmax);
+                        m_run = bmax;
+                    }
+                    float acc0 = 0.f, acc1 = 0.f;
+#pragma unroll
+                    for (int j = 0; j < 32; j += 2) {
+                        acc0 += fast_ex2(l[j] - m_run);
+                        acc1 += fast_ex2(l[j + 1] - m_run);
+                    }
+                    s_run += acc0 + acc1;
+                    // the LIST largest: most blocks hold nothing that beats any lane's current LIST-th value
+                    if (__any_sync(0xffffffffu, bmax > tv[LIST - 1])) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            if (l[j] > tv[LIST - 1]) {              // strict: of equal values the smaller index stays
+                                tv[LIST - 1] = l[j];
+                                ti[LIST - 1] = col0 + j;
+#pragma unroll
+                                for (int q = LIST - 1; q > 0; --q) {
+                                    if (tv[q] > tv[q - 1]) {
+                                        const float fv = tv[q]; tv[q] = tv[q - 1]; tv[q - 1] = fv;
+                                        const int fi = ti[q]; ti[q] = ti[q - 1]; ti[q - 1] = fi;
+                                    }
+                                }
+                            }
+                        }
+                    }
+                }
+            }
+            if (alive && row < p.n) {
+                float w[RECW];
+                w[0] = m_run;
+                w[1] = s_run;
+#pragma unroll
+                for (int j = 0; j < LIST; ++j) { w[2 + j] = tv[j]; w[2 + LIST + j] = __int_as_float(ti[j]); }
+#pragma unroll
+                for (int j = 2 + 2 * LIST; j < RECW; ++j) w[j] = 0.f;
+                float4* dst = reinterpret_cast<float4*>(p.rec + ((size_t)row * 2 + grp) * RECW);
+#pragma unroll
+                for (int j = 0; j < RECW; j += 4) dst[j >> 2] = make_float4(w[j], w[j + 1], w[j + 2], w[j + 3]);
+            }
+        }
+    } else if (warp == AT_PRODUCER) {
+        // =========================== producer warp (TMA) ===========================
+        // Order of the loads = order of use: the tile's A atoms are interleaved with the B stages of its first chunk.  An A
+        // atom of the next tile is loaded as soon as the last chunk's MMAs over that atom have completed, i.e. while the
+        // rest of that chunk still runs.
+        int64_t g = 0;                               // B steps issued
+        int64_t a_tile[4] = {-1, -1, -1, -1};        // last tile whose atom was requested
+        bool ok = true;
+        auto wait0 = [&](uint32_t bar, uint32_t parity) -> bool {
+            uint32_t w = 1;
+            if (lane == 0) w = bar_wait(bar, parity, abort_flag, p.status, false) ? 1u : 0u;
+            return __shfl_sync(0xffffffffu, w, 0) != 0u;
+        };
+        for (int64_t i = 0; i < ntl && ok; ++i) {
+            const int32_t row0 = (int32_t)((blockIdx.x + i * gridDim.x) * AT_POINTS);
+            for (int c = 0; c < NC && ok; ++c) {
+                for (int a = 0; a < n_atoms && ok; ++a) {
+                    if (c == 0) {
+                        if (i > 0 && !wait0(BAR(AB_AEMPTY + a), (uint32_t)((i - 1) & 1))) { ok = false; break; }
+                        if (elect_one()) {
+                            bar_expect_tx(BAR(AB_AFULL + a), 2 * AT_ATOM);
+                            tma_load_3d(smem_u32(smem + ASM_A + a * AT_ATOM), &tm_yhi, 0, row0, a, BAR(AB_AFULL + a));
+                            tma_load_3d(smem_u32(smem + ASM_ALO + a * AT_ATOM), &tm_ylo, 0, row0, a, BAR(AB_AFULL + a));
+                            if (i + 1 < ntl) {       // the planes come from HBM: ask for the next tile's atom now
+                                const int32_t rown = (int32_t)((blockIdx.x + (i + 1) * gridDim.x) * AT_POINTS);
+                                tma_prefetch_3d(&tm_yhi, 0, rown, a);
+                                tma_prefetch_3d(&tm_ylo, 0, rown, a);
+                            }
+                        }
+                        __syncwarp();
+                        a_tile[a] = i;
+                    }
+                    const int st = (int)(g % AT_STAGES);
+                    const int64_t use = g / AT_STAGES;
+                    if (use > 0 && !wait0(BAR(AB_BEMPTY + st), (uint32_t)((use - 1) & 1))) { ok = false; break; }
+                    if (elect_one()) {
+                        const uint32_t dst = smem_u32(smem + ASM_B + st * 2 * AT_ATOM);
+                        bar_expect_tx(BAR(AB_BFULL + st), 2 * AT_ATOM);
+                        tma_load_3d(dst, &tm_phi, 0, c * AT_COMPS, a, BAR(AB_BFULL + st));
+                        tma_load_3d(dst + AT_ATOM, &tm_plo, 0, c * AT_COMPS, a, BAR(AB_BFULL + st));
+                    }
+                    __syncwarp();
+                    ++g;
+                }
+            }
+        }
+        // After an abort nobody may be waiting for the last loads, yet they must have landed before the CTA exits.
+        if (!ok || *abort_flag) {
+            for (int a = 0; a < 4; ++a) {
+                if (a_tile[a] >= 0 && lane == 0) bar_wait(BAR(AB_AFULL + a), (uint32_t)(a_tile[a] & 1), drain_flag, p.status, false);
+                __syncwarp();
+            }
+            for (int64_t h = (g > AT_STAGES ? g - AT_STAGES : 0); h < g; ++h) {
+                if (lane == 0) bar_wait(BAR(AB_BFULL + (int)(h % AT_STAGES)), (uint32_t)((h / AT_STAGES) & 1), drain_flag, p.status, false);
+                __syncwarp();
+            }
+        }
+    } else {
+        // =========================== MMA warp ===========================
+        // The whole warp runs the loop convergently: lane 0 waits and broadcasts, one elected lane issues and commits.
+        const uint32_t idesc = make_idesc(AT_POINTS, AT_COMPS, 0);
+        const uint64_t d_ahi = make_desc(smem_u32(smem + ASM_A), 16, 1024);
+        const uint64_t d_alo = make_desc(smem_u32(smem + ASM_ALO), 16, 1024);
+        const uint64_t d_b = make_desc(smem_u32(smem + ASM_B), 16, 1024);
+        bool alive = true;
+        auto wait_all = [&](uint32_t bar, uint32_t parity) -> bool {
+            uint32_t ok = 1;
+            if (lane == 0) ok = bar_wait(bar, parity, abort_flag, p.status, false) ? 1u : 0u;
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            fence_after();
+            return ok != 0u;
+        };
+        int64_t g = 0;
+        uint32_t cnt[2] = {0u, 0u};
+        for (int64_t i = 0; i < ntl && alive; ++i) {
+            for (int c = 0; c < NC && alive; ++c) {
+                const int b = c & 1;
+                if (cnt[b] > 0 && !wait_all(BAR(AB_LEMPTY + b), (cnt[b] - 1) & 1u)) { alive = false; break; }
+                ++cnt[b];
+                const uint32_t d = tmem + b * AT_COMPS;
+                for (int a = 0; a < n_atoms; ++a) {
+                    if (c == 0 && !wait_all(BAR(AB_AFULL + a), (uint32_t)(i & 1))) { alive = false; break; }
+                    const int st = (int)(g % AT_STAGES);
+                    if (!wait_all(BAR(AB_BFULL + st), (uint32_t)((g / AT_STAGES) & 1))) { alive = false; break; }
+                    if (elect_one()) {
+                        const int kk = (p.n_ks - 4 * a < 4) ? (p.n_ks - 4 * a) : 4;          // k-steps of this atom
+                        const uint64_t ah = d_ahi + ((a * AT_ATOM) >> 4), al = d_alo + ((a * AT_ATOM) >> 4);
+                        const uint64_t bh = d_b + ((st * 2 * AT_ATOM) >> 4), bl = bh + (AT_ATOM >> 4);
+                        // the two small cross products first, then the leading one (as in the E-step of the tile kernel)
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            if (j < kk) mma_ss(d, ah + ((j * 32) >> 4), bl + ((j * 32) >> 4), idesc, (a > 0 || j > 0) ? 1u : 0u);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            if (j < kk) mma_ss(d, al + ((j * 32) >> 4), bh + ((j * 32) >> 4), idesc, 1u);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            if (j < kk) mma_ss(d, ah + ((j * 32) >> 4), bh + ((j * 32) >> 4), idesc, 1u);
+                        mma_commit(BAR(AB_BEMPTY + st));
+                        if (c == NC - 1) mma_commit(BAR(AB_AEMPTY + a));
+                        if (a == n_atoms - 1) mma_commit(BAR(AB_LFULL + b));
+                    }
+                    __syncwarp();
+                    ++g;
+                }
+            }
+        }
+        // drain: every MMA issued by this warp has completed before TMEM is released
+        if (elect_one()) mma_commit(BAR(AB_FINAL));
+        __syncwarp();
+        if (lane == 0) bar_wait(BAR(AB_FINAL), 0, drain_flag, p.status, false);
+        __syncwarp();
+        fence_after();
+    }
+
+    fence_before();
+    __syncthreads();
+    if (warp == AT_MMA) {
+        fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(256) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------------------
+// Exact log2 z of (point, component) pairs by direct differences in fp32, one warp per point: lane l holds the
+// dimensions l, l + 32, l + 64, l + 96 of the point.
+struct PointRow {
+    float x[4];
+    __device__ __forceinline__ void load(const float* __restrict__ xr, int D, int lane) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) x[j] = (lane + 32 * j < D) ? __ldg(xr + lane + 32 * j) : 0.f;
+    }
+    // sum_d w (x - mu)^2 and, with MAG, sum_d w (|x| + |mu|)^2 (the size of the terms the expanded form adds up)
+    template <bool MAG>
+    __device__ __forceinline__ float quad(const float* __restrict__ mr, const float* __restrict__ wr, int D, int lane, float& mag) const {
+        float q = 0.f, t = 0.f;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int d = lane + 32 * j;
+            if (d < D) {
+                const float mu = __ldg(mr + d), w = __ldg(wr + d);
+                const float diff = x[j] - mu;
+                q = fmaf(diff * diff, w, q);
+                if (MAG) { const float a = fabsf(x[j]) + fabsf(mu); t = fmaf(a * a, w, t); }
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            q += __shfl_xor_sync(0xffffffffu, q, o);
+            if (MAG) t += __shfl_xor_sync(0xffffffffu, t, o);
+        }
+        mag = t;
+        return q;
+    }
+};
+
+template <int LIST>
+__global__ void __launch_bounds__(256)
+assign_refine_kernel(const float* __restrict__ rec, const float* __restrict__ X, int64_t n, int D, int K,
+                     const float* __restrict__ mu, const float* __restrict__ w2, const float* __restrict__ c2,
+                     const int* __restrict__ flags, const int* __restrict__ ill_list, int m, int32_t* __restrict__ idx_out,
+                     float* __restrict__ resp_out) {
+    if (flags[3] != 0) return;
+    constexpr int RECW = assign_recw(LIST);
+    constexpr int C = LIST - 1;                                  // candidates recomputed exactly
+    const float e_launch = __int_as_float(flags[1]);             // error bound of the approximate logits from the parameters
+    const int n_ill = flags[2];                                  // ill-conditioned components (<= 32): always evaluated exactly
+    const int lane = threadIdx.x & 31;
+    const int ill_k = (lane < n_ill) ? __ldg(ill_list + lane) : -1;      // lane t keeps ill-conditioned component t
+    const int64_t warp0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    const float NEG = -CUDART_INF_F;
+    for (int64_t row = warp0; row < n; row += nwarps) {
+        const float* r0 = rec + (size_t)row * 2 * RECW;
+        float av = NEG;
+        int ai = -1;
+        if (lane < 2 * LIST) {
+            const int h = lane / LIST, j = lane - h * LIST;
+            av = __ldg(r0 + h * RECW + 2 + j);
+            ai = __float_as_int(__ldg(r0 + h * RECW + 2 + LIST + j));
+        }
+        const float m0 = __ldg(r0), s0 = __ldg(r0 + 1), m1 = __ldg(r0 + RECW), s1 = __ldg(r0 + RECW + 1);
+        // rank inside the union of the two lists: descending approximate value, ties to the smaller index
+        int rank = 0;
+#pragma unroll
+        for (int t = 0; t < 2 * LIST; ++t) {
+            const float ov = __shfl_sync(0xffffffffu, av, t);
+            const int oi = __shfl_sync(0xffffffffu, ai, t);
+            if (t != lane && oi >= 0 && (ai < 0 || ov > av || (ov == av && oi < ai))) ++rank;
+        }
+        const int nvalid = __popc(__ballot_sync(0xffffffffu, ai >= 0));
+        const int nc = nvalid < C ? nvalid : C;
+        PointRow pr;
+        pr.load(X + row * D, D, lane);
+        // exact values of the candidates: lane r keeps candidate r (in the order of the approximate values)
+        float ev = NEG, ea = NEG, tmax = 0.f;
+        int ek = -1;
+        for (int r = 0; r < nc; ++r) {
+            const int src = __ffs(__ballot_sync(0xffffffffu, ai >= 0 && rank == r)) - 1;
+            const int k = __shfl_sync(0xffffffffu, ai, src);
+            const float a = __shfl_sync(0xffffffffu, av, src);
+            float mag;
+            const float q = pr.quad<true>(mu + (size_t)k * D, w2 + (size_t)k * D, D, lane, mag);
+            const float e = __ldg(c2 + k) - q;
+            tmax = fmaxf(tmax, mag);
+            if (lane == r) { ev = e; ea = a; ek = k; }
+        }
+        // ... and of the ill-conditioned components, which the approximate pass left out (constant -inf there)
+        float iv = NEG;
+        for (int t = 0; t < n_ill; ++t) {
+            const int k = __shfl_sync(0xffffffffu, ill_k, t);
+            float mag;
+            const float q = pr.quad<false>(mu + (size_t)k * D, w2 + (size_t)k * D, D, lane, mag);
+            const float e = __ldg(c2 + k) - q;
+            if (lane == t) iv = e;
+        }
+        const int ik = (iv > NEG) ? ill_k : -1;                   // an ill-conditioned component of zero weight counts as absent here
+        float nxt = NEG;                                          // best approximate value outside the candidates
+        if (nvalid > C) {
+            const int src = __ffs(__ballot_sync(0xffffffffu, ai >= 0 && rank == C)) - 1;
+            nxt = __shfl_sync(0xffffffffu, av, src);
+        }
+        // order of all exactly known values (a lane holds up to two: a candidate and an ill-conditioned component)
+        int erank = 0, irank = 0;
+        const int span = (n_ill > 0) ? 32 : C;
+        for (int t = 0; t < span; ++t) {
+            const float ov = __shfl_sync(0xffffffffu, ev, t);
+            const int ok = __shfl_sync(0xffffffffu, ek, t);
+            if (ok >= 0) {
+                if (t != lane && (ek < 0 || ov > ev || (ov == ev && ok < ek))) ++erank;
+                if (ik < 0 || ov > iv || (ov == iv && ok < ik)) ++irank;
+            }
+            if (n_ill > 0) {
+                const float pv = __shfl_sync(0xffffffffu, iv, t);
+                const int pk = __shfl_sync(0xffffffffu, ik, t);
+                if (pk >= 0) {
+                    if (ek < 0 || pv > ev || (pv == ev && pk < ek)) ++erank;
+                    if (t != lane && (ik < 0 || pv > iv || (pv == iv && pk < ik))) ++irank;
+                }
+            }
+        }
+        const int nexact = __popc(__ballot_sync(0xffffffffu, ek >= 0)) + __popc(__ballot_sync(0xffffffffu, ik >= 0));
+        float e_m = NEG;                                          // m-th largest exact value
+        {
+            const unsigned b1 = __ballot_sync(0xffffffffu, ek >= 0 && erank == m - 1);
+            const unsigned b2 = __ballot_sync(0xffffffffu, ik >= 0 && irank == m - 1);
+            if (b1) e_m = __shfl_sync(0xffffffffu, ev, __ffs(b1) - 1);
+            else if (b2) e_m = __shfl_sync(0xffffffffu, iv, __ffs(b2) - 1);
+        }
+        // Error bound of an approximate logit: from the parameters (8 x the estimate, over the components that take part
+        // in the approximate pass) and from this point (8 x 2^-22 x the summed magnitude of the terms, largest over the
+        // candidates).
+        const float ebound = e_launch + 1.9073486e-06f * tmax;
+        bool certain = nexact >= m && (nvalid <= C || e_m > nxt + ebound);
+        float M = fmaxf(m0, m1), S = 0.f;
+        if (certain) {
+            float emax = fmaxf(ev, iv);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) emax = fmaxf(emax, __shfl_xor_sync(0xffffffffu, emax, o));
+            M = fmaxf(M, emax);
+            // log-sum-exp: the approximate total with the candidates' approximate terms replaced by the exact ones, plus
+            // the ill-conditioned components
+            float corr = (ek >= 0) ? (fast_ex2(ev - M) - fast_ex2(ea - M)) : 0.f;
+            if (ik >= 0) corr += fast_ex2(iv - M);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) corr += __shfl_xor_sync(0xffffffffu, corr, o);
+            S = s0 * fast_ex2(m0 - M) + s1 * fast_ex2(m1 - M) + corr;
+            if (!(S > 0.f) || !(S < CUDART_INF_F)) certain = false;
+        }
+        if (certain) {
+            if (ek >= 0 && erank < m) {
+                idx_out[row * m + erank] = ek;
+                resp_out[row * m + erank] = __fdividef(fast_ex2(ev - M), S);
+            }
+            if (ik >= 0 && irank < m) {
+                idx_out[row * m + irank] = ik;
+                resp_out[row * m + irank] = __fdividef(fast_ex2(iv - M), S);
+            }
+            continue;
+        }
+        // ---- not certain (near ties, exact ties, too few finite candidates): all K components exactly ----
+        float tv[GMM_MAX_TOPM];
+        int ti[GMM_MAX_TOPM];
+#pragma unroll
+        for (int j = 0; j < GMM_MAX_TOPM; ++j) { tv[j] = NEG; ti[j] = -1; }
+        float Mx = NEG, Sx = 0.f;
+        for (int k = 0; k < K; ++k) {
+            float mag;
+            const float q = pr.quad<false>(mu + (size_t)k * D, w2 + (size_t)k * D, D, lane, mag);
+            const float e = __ldg(c2 + k) - q;
+            if (e > Mx) { Sx = Sx * fast_ex2(Mx - e) + 1.f; Mx = e; }        // (Mx = -inf: Sx is 0, and 0 * 2^-inf = 0)
+            else if (e > NEG) Sx += fast_ex2(e - Mx);
+            // the GMM_MAX_TOPM largest (their first m are the answer): descending order, equal values keep the smaller index
+            // first, -inf values fill a list that is not full yet
+            if (ti[GMM_MAX_TOPM - 1] < 0 || e > tv[GMM_MAX_TOPM - 1]) {
+                tv[GMM_MAX_TOPM - 1] = e;
+                ti[GMM_MAX_TOPM - 1] = k;
+#pragma unroll
+                for (int j = GMM_MAX_TOPM - 1; j > 0; --j) {
+                    if (ti[j] >= 0 && (ti[j - 1] < 0 || tv[j] > tv[j - 1])) {
+                        const float fv = tv[j]; tv[j] = tv[j - 1]; tv[j - 1] = fv;
+                        const int fi = ti[j]; ti[j] = ti[j - 1]; ti[j - 1] = fi;
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < GMM_MAX_TOPM; ++j) {
+            if (j < m && lane == 0) {
+                idx_out[row * m + j] = ti[j] >= 0 ? ti[j] : 0;
+                resp_out[row * m + j] = (ti[j] >= 0 && tv[j] > NEG && Sx > 0.f) ? __fdividef(fast_ex2(tv[j] - Mx), Sx) : 0.f;
+            }
+        }
+    }
+}
+
+template <int LIST>
+cudaError_t launch_assign_t(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu, const float* w2,
+                            const float* c2, const TcBuffers& tb, float* rec, int m, int32_t* idx, float* resp, int* status) {
+    const TcPlan pl = tc_plan(D, K, 148);
+    AssignParams p;
+    p.n = n; p.n_chunks = pl.CL; p.n_ks = pl.n_ks;
+    p.tkck = reinterpret_cast<const float2*>(tb.tkck);
+    p.rec = rec; p.status = status; p.gate = tb.flags + 3;
+    const int64_t rows_padded = (n + TC_BN - 1) / TC_BN * TC_BN;       // what launch_transform_tc wrote
+    CUtensorMap tm_yhi, tm_ylo, tm_phi, tm_plo;
+    cudaError_t e = tc_make_plane_map(&tm_yhi, tb.y_hi, rows_padded, AT_POINTS, 1);
+    if (e != cudaSuccess) return e;
+    e = tc_make_plane_map(&tm_ylo, tb.y_lo, rows_padded, AT_POINTS, 1);
+    if (e != cudaSuccess) return e;
+    e = tc_make_plane_map(&tm_phi, tb.p_hi_rm, pl.Kpad, AT_COMPS, 1);
+    if (e != cudaSuccess) return e;
+    e = tc_make_plane_map(&tm_plo, tb.p_lo_rm, pl.Kpad, AT_COMPS, 1);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(assign_tc_kernel<LIST>, cudaFuncAttributeMaxDynamicSharedMemorySize, ASM_BYTES);
+    if (e != cudaSuccess) return e;
+    int dev = 0, sms = 0;
+    e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    const int64_t ntiles = (n + AT_POINTS - 1) / AT_POINTS;
+    const unsigned grid = (unsigned)(ntiles < sms ? ntiles : sms);          // persistent: one CTA per SM
+    assign_tc_kernel<LIST><<<grid, AT_THREADS, ASM_BYTES, s>>>(p, tm_yhi, tm_ylo, tm_phi, tm_plo);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const int64_t warps_wanted = n < (int64_t)sms * 64 ? n : (int64_t)sms * 64;      // 8 CTAs of 8 warps per SM
+    const unsigned rgrid = (unsigned)((warps_wanted + 7) / 8);
+    assign_refine_kernel<LIST><<<rgrid, 256, 0, s>>>(rec, X, n, D, K, mu, w2, c2, tb.flags, tb.ill_list, m, idx, resp);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+size_t assign_tc_record_bytes(int m) { return (size_t)2 * (m <= 4 ? assign_recw(8) : assign_recw(12)) * sizeof(float); }
+
+cudaError_t launch_assign_tc(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu, const float* w2,
+                             const float* c2, const TcBuffers& tb, float* rec, int m, int32_t* idx, float* resp, int* status) {
+    if (n < 1 || n > TC_YPOINTS || m < 1 || m > GMM_MAX_TOPM) return cudaErrorInvalidValue;
+    if (m <= 4) return launch_assign_t<8>(s, X, n, D, K, mu, w2, c2, tb, rec, m, idx, resp, status);
+    return launch_assign_t<12>(s, X, n, D, K, mu, w2, c2, tb, rec, m, idx, resp, status);
+}
+
+}  // namespace fg

@@ -155,8 +155,11 @@ template <int M, typename ACC>
 __global__ void __launch_bounds__(NTHREADS)
 lse_kernel(const float* __restrict__ X, int64_t n, int D, int K, const float* __restrict__ mu,
            const float* __restrict__ w2, const double* __restrict__ c2, double* __restrict__ logZ2,
-           double* __restrict__ llpart, int m_out, int32_t* __restrict__ idx_out, float* __restrict__ resp_out) {
+           double* __restrict__ llpart, int m_out, int32_t* __restrict__ idx_out, float* __restrict__ resp_out,
+           const int* __restrict__ run_if) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
+    // run_if: the launch does nothing unless run_if[0] != 0 (the tensor-core assignment covers the other case)
+    if (run_if && run_if[0] == 0) return;
     TileSmem& sm = *reinterpret_cast<TileSmem*>(smem_raw);
     __shared__ double ll_s[TP];
     const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
@@ -583,37 +586,37 @@ cudaError_t launch_lse_fp32(cudaStream_t s, const float* X, int64_t n, int D, in
                             const float* w2, const double* c2d, double* logZ2, double* llpart) {
     const unsigned blocks = (unsigned)((n + TP - 1) / TP);
     if (fp32_high_precision(D))
-        lse_kernel<0, double><<<blocks, NTHREADS, sizeof(TileSmem), s>>>(X, n, D, K, mu, w2, c2d, logZ2, llpart, 0, nullptr, nullptr);
+        lse_kernel<0, double><<<blocks, NTHREADS, sizeof(TileSmem), s>>>(X, n, D, K, mu, w2, c2d, logZ2, llpart, 0, nullptr, nullptr, nullptr);
     else
-        lse_kernel<0, float><<<blocks, NTHREADS, sizeof(TileSmem), s>>>(X, n, D, K, mu, w2, c2d, logZ2, llpart, 0, nullptr, nullptr);
+        lse_kernel<0, float><<<blocks, NTHREADS, sizeof(TileSmem), s>>>(X, n, D, K, mu, w2, c2d, logZ2, llpart, 0, nullptr, nullptr, nullptr);
     return cudaGetLastError();
 }
 
 template <int M, typename ACC>
 static cudaError_t launch_topm_t(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu,
-                                 const float* w2, const double* c2d, int m, int32_t* idx, float* resp) {
+                                 const float* w2, const double* c2d, int m, int32_t* idx, float* resp, const int* run_if) {
     size_t smem = sizeof(TileSmem);
     const size_t need = (size_t)TP * 16 * M * (sizeof(ACC) + 4);
     if (need > smem) smem = need;
     cudaError_t e = cudaFuncSetAttribute(lse_kernel<M, ACC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     const unsigned blocks = (unsigned)((n + TP - 1) / TP);
-    lse_kernel<M, ACC><<<blocks, NTHREADS, smem, s>>>(X, n, D, K, mu, w2, c2d, nullptr, nullptr, m, idx, resp);
+    lse_kernel<M, ACC><<<blocks, NTHREADS, smem, s>>>(X, n, D, K, mu, w2, c2d, nullptr, nullptr, m, idx, resp, run_if);
     return cudaGetLastError();
 }
 
 cudaError_t launch_topm_fp32(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu,
-                             const float* w2, const double* c2d, int m, int32_t* idx, float* resp) {
+                             const float* w2, const double* c2d, int m, int32_t* idx, float* resp, const int* run_if) {
     if (fp32_high_precision(D)) {
-        if (m <= 1) return launch_topm_t<1, double>(s, X, n, D, K, mu, w2, c2d, m, idx, resp);
-        if (m <= 2) return launch_topm_t<2, double>(s, X, n, D, K, mu, w2, c2d, m, idx, resp);
-        if (m <= 4) return launch_topm_t<4, double>(s, X, n, D, K, mu, w2, c2d, m, idx, resp);
-        return launch_topm_t<8, double>(s, X, n, D, K, mu, w2, c2d, m, idx, resp);
+        if (m <= 1) return launch_topm_t<1, double>(s, X, n, D, K, mu, w2, c2d, m, idx, resp, run_if);
+        if (m <= 2) return launch_topm_t<2, double>(s, X, n, D, K, mu, w2, c2d, m, idx, resp, run_if);
+        if (m <= 4) return launch_topm_t<4, double>(s, X, n, D, K, mu, w2, c2d, m, idx, resp, run_if);
+        return launch_topm_t<8, double>(s, X, n, D, K, mu, w2, c2d, m, idx, resp, run_if);
     }
-    if (m <= 1) return launch_topm_t<1, float>(s, X, n, D, K, mu, w2, c2d, m, idx, resp);
-    if (m <= 2) return launch_topm_t<2, float>(s, X, n, D, K, mu, w2, c2d, m, idx, resp);
-    if (m <= 4) return launch_topm_t<4, float>(s, X, n, D, K, mu, w2, c2d, m, idx, resp);
-    return launch_topm_t<8, float>(s, X, n, D, K, mu, w2, c2d, m, idx, resp);
+    if (m <= 1) return launch_topm_t<1, float>(s, X, n, D, K, mu, w2, c2d, m, idx, resp, run_if);
+    if (m <= 2) return launch_topm_t<2, float>(s, X, n, D, K, mu, w2, c2d, m, idx, resp, run_if);
+    if (m <= 4) return launch_topm_t<4, float>(s, X, n, D, K, mu, w2, c2d, m, idx, resp, run_if);
+    return launch_topm_t<8, float>(s, X, n, D, K, mu, w2, c2d, m, idx, resp, run_if);
 }
 
 cudaError_t launch_mstep_fp32(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu,

@@ -37,6 +37,15 @@
 #include <math_constants.h>
 
 namespace fg {
+namespace {
+// Wall-clock limit of every device-side wait, in ns (2 s; a test of the time-out path shortens it).
+__constant__ unsigned long long c_wait_limit_ns = 2000000000ull;
+}  // namespace
+}  // namespace fg
+#define TC_WAIT_LIMIT_NS c_wait_limit_ns
+#include "tc_prims.cuh"
+
+namespace fg {
 
 namespace {
 
@@ -45,9 +54,7 @@ constexpr int NTHREADS = 320;          // 8 softmax warps, 1 producer warp, 1 MM
 constexpr int MMA_WARP = 9;
 constexpr int PRODUCER_WARP = 8;
 constexpr float RSCALE = TC_RSCALE;
-// Wall-clock limit of every device-side wait, in ns (2 s; a test of the time-out path shortens it).
-__constant__ unsigned long long c_wait_limit_ns = 2000000000ull;
-#define WAIT_LIMIT_NS c_wait_limit_ns
+#define WAIT_LIMIT_NS TC_WAIT_LIMIT_NS
 constexpr float ILL_MARGIN = 40.f;     // log2 units: a logit more than this below the best one is negligible (2^-40)
 
 // shared memory map (offsets from a 1024-byte aligned base)
@@ -77,89 +84,6 @@ enum { B_YFULL0 = 0, B_YFULL1, B_YEMPTY0, B_YEMPTY1, B_LFULL0, B_LFULL1, B_RREAD
 #define TRACE(ev, tile)
 #endif
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ unsigned long long gtime() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-
-__device__ __forceinline__ float fast_ex2(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-
-__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-    uint64_t d = 0;
-    d |= (uint64_t)((saddr >> 4) & 0x3FFF);
-    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
-    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
-    d |= (uint64_t)1 << 46;       // descriptor version
-    d |= (uint64_t)2 << 61;       // 128-byte swizzle
-    return d;
-}
-
-__device__ __forceinline__ uint32_t make_idesc(int M, int N, int b_mn_major) {
-    uint32_t d = 0;
-    d |= 1u << 4;                                // D: f32
-    d |= (uint32_t)b_mn_major << 16;             // A, B: f16; A K-major
-    d |= (uint32_t)(N >> 3) << 17;
-    d |= (uint32_t)(M >> 4) << 24;
-    return d;
-}
-
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t acc) {
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}\n"
-                 ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(acc) : "memory");
-}
-__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b, uint32_t idesc, uint32_t acc) {
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                 "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}\n"
-                 ::"r"(d_tmem), "r"(a_tmem), "l"(b), "r"(idesc), "r"(acc) : "memory");
-}
-__device__ __forceinline__ void mma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-// One lane of a converged warp (all 32 lanes must call it together).
-__device__ __forceinline__ bool elect_one() {
-    uint32_t pred;
-    asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xffffffff;\n\tselp.u32 %0, 1, 0, P;\n\t}\n" : "=r"(pred)::"memory");
-    return pred != 0u;
-}
-
-__device__ __forceinline__ void bar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void bar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void bar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-// One tile (box fixed by the tensor map) from global to shared memory; completion is counted in bytes on `bar`.
-// x = innermost coordinate in elements (always 0 here), y = first row, z = first atom.
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, int32_t x, int32_t y, int32_t z, uint32_t bar) {
-    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-                 ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
-}
-// Asks for one tile of a tensor to be brought into L2 (no destination, no completion).
-__device__ __forceinline__ void tma_prefetch_3d(const CUtensorMap* tm, int32_t x, int32_t y, int32_t z) {
-    asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];"
-                 ::"l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(z) : "memory");
-}
-// Non-blocking test of an mbarrier phase.
-__device__ __forceinline__ bool bar_test(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
-                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0u;
-}
 // ---- exchange between the CTAs of a group through global memory (L2).  A slot is two 64-bit words {value, tag}: each
 //      word is written and read as one unit, so a reader that sees the expected tag in both words has both values.
 //      Slots form a ring of 4 per (group, source CTA): a CTA writes tile i+4 only after it has finished tile i+2, which
@@ -172,30 +96,6 @@ __device__ __forceinline__ void xslot_write(XSlot* q, float a, float b, uint32_t
 __device__ __forceinline__ void xslot_load(const XSlot* q, uint32_t (&v)[4]) {
     asm volatile("ld.relaxed.gpu.global.v4.b32 {%0, %1, %2, %3}, [%4];"
                  : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]) : "l"(q) : "memory");
-}
-// Bounded wait on an mbarrier phase.  Returns false on abort/timeout (and raises the abort flag).
-__device__ __forceinline__ bool bar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, bool cluster_scope) {
-    unsigned long long t0 = 0;
-    for (int it = 0;; ++it) {
-        uint32_t ok;
-        if (cluster_scope)
-            asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
-                         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-        else
-            asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
-                         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-        if (ok) return true;
-        if (*abort_flag) return false;
-        if ((it & 63) == 63) {
-            const unsigned long long now = gtime();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > WAIT_LIMIT_NS) {
-                *abort_flag = 1;
-                atomicOr(status, ST_TIMEOUT);
-                return false;
-            }
-        }
-    }
 }
 
 // Bounded poll of the CL slots of one point (stride 64 slots between source CTAs): all outstanding loads are issued
@@ -234,40 +134,6 @@ __device__ __forceinline__ bool xslot_wait_all(const XSlot* q, int CL, uint32_t 
     }
 }
 
-__device__ __forceinline__ void named_bar_sync(int id, int count) {
-    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
-}
-
-// ---- TMEM load / store helpers (32 lanes x 32 columns per call; thread = lane) ----
-__device__ __forceinline__ void tmem_ld32(uint32_t addr, uint32_t (&v)[32]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
-          "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
-          "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-        : "r"(addr) : "memory");
-}
-__device__ __forceinline__ void tmem_st32(uint32_t addr, const uint32_t (&v)[32]) {
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-        "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
-        ::"r"(addr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]),
-          "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]), "r"(v[16]), "r"(v[17]),
-          "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]), "r"(v[24]), "r"(v[25]), "r"(v[26]),
-          "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
-        : "memory");
-}
-__device__ __forceinline__ void tmem_st16(uint32_t addr, const uint32_t (&v)[16]) {
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
-        ::"r"(addr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]),
-          "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
-        : "memory");
-}
-__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 // ---- warp reduce-scatter butterflies over 64 per-thread values: afterwards lane l holds the reduction (over the
 //      32 lanes) for points 2l and 2l+1.  62 shuffles instead of 64 x 5.
@@ -1161,7 +1027,8 @@ __global__ void __launch_bounds__(128) tc_prepare_kernel(int D, int K, const flo
                                                          uint32_t* __restrict__ phi_img,
                                                          unsigned char* __restrict__ plo_img, float* __restrict__ tk,
                                                          float* __restrict__ ck, float* __restrict__ illb, float cond_limit,
-                                                         int* __restrict__ flags) {
+                                                         int* __restrict__ flags, uint32_t* __restrict__ phi_rm,
+                                                         uint32_t* __restrict__ plo_rm, float2* __restrict__ tkck) {
     const int k = blockIdx.x, d = threadIdx.x;
     const int slice = k >> 7, row = k & 127;
     __shared__ double red_max[128], red_c[128], red_cond[128], red_k[128];
@@ -1207,6 +1074,10 @@ __global__ void __launch_bounds__(128) tc_prepare_kernel(int D, int K, const flo
     // P_hi image: [slice][row][128] packed pairs (even column in the low half)
     phi_img[((size_t)slice * 128 + row) * 128 + d] =
         (uint32_t)__half_as_ushort(hi_s[2 * d]) | ((uint32_t)__half_as_ushort(hi_s[2 * d + 1]) << 16);
+    // The same coefficients as two plain row-major planes [component][256 halves] (the B operand of the assignment kernel,
+    // fetched by TMA, which applies the swizzle itself)
+    phi_rm[(size_t)k * 128 + d] = (uint32_t)__half_as_ushort(hi_s[2 * d]) | ((uint32_t)__half_as_ushort(hi_s[2 * d + 1]) << 16);
+    plo_rm[(size_t)k * 128 + d] = (uint32_t)__half_as_ushort(lo_s[2 * d]) | ((uint32_t)__half_as_ushort(lo_s[2 * d + 1]) << 16);
     // P_lo image: SW128 K-major, atoms of 64 columns, 128 rows
     for (int c = d; c < 256; c += 128) {
         const int atom = c >> 6, cc = c & 63;
@@ -1221,6 +1092,7 @@ __global__ void __launch_bounds__(128) tc_prepare_kernel(int D, int K, const flo
         }
         tk[k] = (float)t;
         ck[k] = c;
+
         // conditioning estimate of the expanded form: 2^-22 sum_d w2 * 3 (mu^2 + 9 var) ~ absolute log2 error bound
         const double cond = red_cond[0] * 2.384185791015625e-07;
         float margin = 0.f;
@@ -1229,7 +1101,34 @@ __global__ void __launch_bounds__(128) tc_prepare_kernel(int D, int K, const flo
             atomicOr(flags, 1);
         }
         illb[k] = margin;
+        // For the assignment kernels: an ill-conditioned component takes no part in the approximate selection (constant
+        // -inf; it is evaluated exactly for every point instead), and flags[1] = the largest error bound (8 x the estimate)
+        // over the other components, as the bits of a non-negative float (their integer order is the order of the floats).
+        tkck[k] = make_float2((float)t, margin > 0.f ? -CUDART_INF_F : c);
+        if (k < K && margin == 0.f) {
+            const float eb = (float)fmin(8.0 * cond, 1e30);
+            if (eb > 0.f) atomicMax(flags + 1, __float_as_int(eb));
+        }
     }
+}
+
+// Ascending list of the ill-conditioned components (illb > 0): flags[2] = their number, flags[3] = 1 when there are more
+// than TC_MAX_ILL of them (the assignment then runs on the FP32 kernels).  One block of 1024 threads, Kpad <= 1024.
+__global__ void __launch_bounds__(1024) tc_ill_list_kernel(int Kpad, const float* __restrict__ illb, int* __restrict__ ill_list,
+                                                           int* __restrict__ flags) {
+    __shared__ int wcount[32];
+    const int k = threadIdx.x, lane = k & 31, w = k >> 5;
+    const bool is = k < Kpad && illb[k] > 0.f;
+    const unsigned b = __ballot_sync(0xffffffffu, is);
+    if (lane == 0) wcount[w] = __popc(b);
+    __syncthreads();
+    int before = 0, total = 0;
+    for (int j = 0; j < 32; ++j) {
+        if (j < w) before += wcount[j];
+        total += wcount[j];
+    }
+    if (is) ill_list[before + __popc(b & ((1u << lane) - 1u))] = k;
+    if (k == 0) { flags[2] = total; flags[3] = total > TC_MAX_ILL ? 1 : 0; }
 }
 
 // stats (+)= sum over Q cluster partials (float64, fixed order), undoing the responsibility scale, the per-dimension
@@ -1310,6 +1209,7 @@ size_t tc_scratch_bytes(int D, int K) {
     b += (size_t)pl.CL * 128 * 128 * 4;                    // P_hi image
     b += (size_t)pl.CL * 65536;                            // P_lo image
     b += (size_t)pl.Kpad * 4 * 2 + 512;                    // t_k, c_k, s_d
+    b += (size_t)pl.Kpad * (512 * 2 + 8 + 4);              // row-major P planes, (t_k, c_k) pairs, list of ill-conditioned components
     b += (size_t)pl.Q * pl.Kpad * TC_PCOLS * 8;            // float64 partials
     b += (size_t)pl.Q * 16;
     b += 5 * (size_t)pl.Q * 4 * pl.CL * 64 * 16;           // exchange slots
@@ -1318,15 +1218,20 @@ size_t tc_scratch_bytes(int D, int K) {
 }
 
 cudaError_t launch_prepare_tc(cudaStream_t s, int D, int K, const float* pi, const float* mu, const float* var,
-                              const TcBuffers& tb, float cond_limit, int* status) {
+                              const TcBuffers& tb, float cond_limit, int* status, bool ill_list) {
     const TcPlan pl = tc_plan(D, K, 148);
     (void)status;
-    cudaError_t e0 = cudaMemsetAsync(tb.flags, 0, sizeof(int), s);
+    cudaError_t e0 = cudaMemsetAsync(tb.flags, 0, 4 * sizeof(int), s);
     if (e0 != cudaSuccess) return e0;
     tc_scale_kernel<<<128, 128, 0, s>>>(D, K, pi, mu, var, tb.sd, tb.kap);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    tc_prepare_kernel<<<pl.Kpad, 128, 0, s>>>(D, K, pi, mu, var, tb.sd, tb.kap, tb.phi_img, tb.plo_img, tb.tk, tb.ck, tb.illb, cond_limit, tb.flags);
+    tc_prepare_kernel<<<pl.Kpad, 128, 0, s>>>(D, K, pi, mu, var, tb.sd, tb.kap, tb.phi_img, tb.plo_img, tb.tk, tb.ck, tb.illb, cond_limit, tb.flags,
+                                                  reinterpret_cast<uint32_t*>(tb.p_hi_rm), reinterpret_cast<uint32_t*>(tb.p_lo_rm),
+                                                  reinterpret_cast<float2*>(tb.tkck));
+    e = cudaGetLastError();
+    if (e != cudaSuccess || !ill_list) return e;
+    tc_ill_list_kernel<<<1, 1024, 0, s>>>(pl.Kpad, tb.illb, tb.ill_list, tb.flags);
     return cudaGetLastError();
 }
 
@@ -1340,13 +1245,12 @@ cudaError_t launch_transform_tc(cudaStream_t s, const float* X, int64_t n, int D
     return cudaGetLastError();
 }
 
-namespace {
 // A plane [rows][256 halves] seen as a 3-D tensor (x = 64 halves of an atom's row, y = row, z = atom): a box of
-// (64, 64 points, n_atoms) lands in shared memory as [atom][point][128 bytes], each 128-byte row swizzled.
-cudaError_t make_plane_map(CUtensorMap* tm, void* base, int64_t rows, int n_atoms) {
+// (64, box_rows, box_atoms) lands in shared memory as [atom][row][128 bytes], each 128-byte row swizzled.
+cudaError_t tc_make_plane_map(CUtensorMap* tm, void* base, int64_t rows, int box_rows, int box_atoms) {
     const cuuint64_t dims[3] = {64, (cuuint64_t)rows, 4};
     const cuuint64_t strides[2] = {512, 128};                 // bytes between rows, between atoms
-    const cuuint32_t box[3] = {64, (cuuint32_t)TC_BN, (cuuint32_t)n_atoms};
+    const cuuint32_t box[3] = {64, (cuuint32_t)box_rows, (cuuint32_t)box_atoms};
     const cuuint32_t estr[3] = {1, 1, 1};
     // The encoder lives in the driver library; it is looked up at run time so that this library has no load-time
     // dependency on the driver (it must load, e.g. for symbol checks, on a machine without one).
@@ -1367,7 +1271,6 @@ cudaError_t make_plane_map(CUtensorMap* tm, void* base, int64_t rows, int n_atom
                               CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
-}  // namespace
 
 cudaError_t launch_em_tc(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu, const float* w2,
                          const float* c2, const TcBuffers& tb, int Q, int flush_tiles, int* status) {
@@ -1417,9 +1320,9 @@ cudaError_t launch_em_tc(cudaStream_t s, const float* X, int64_t n, int D, int K
     const int64_t rows_padded = (n + TC_BN - 1) / TC_BN * TC_BN;       // launch_transform_tc wrote zeros beyond n
     CUtensorMap tm_hi, tm_lo;
     const int n_atoms = (pl.n_ks + 3) / 4;
-    e = make_plane_map(&tm_hi, tb.y_hi, rows_padded, n_atoms);
+    e = tc_make_plane_map(&tm_hi, tb.y_hi, rows_padded, TC_BN, n_atoms);
     if (e != cudaSuccess) return e;
-    e = make_plane_map(&tm_lo, tb.y_lo, rows_padded, n_atoms);
+    e = tc_make_plane_map(&tm_lo, tb.y_lo, rows_padded, TC_BN, n_atoms);
     if (e != cudaSuccess) return e;
     return cudaLaunchKernelEx(&cfg, em_tc_kernel, p, tm_hi, tm_lo);
 }

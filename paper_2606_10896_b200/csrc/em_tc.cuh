@@ -1,5 +1,6 @@
 // Declarations of the tensor-core path (internal).
 #pragma once
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 #include <stddef.h>
@@ -10,6 +11,7 @@ constexpr int TC_BN = 64;            // points per tile
 constexpr int TC_FLUSH = 64;         // tiles between flushes of the TMEM accumulators into float64 partials (even)
 constexpr float TC_RSCALE = 4096.f;  // responsibilities are scaled by this power of two before the fp16 split
 constexpr int TC_PCOLS = 258;        // columns of a partial row: 256 statistics columns + N_k of each softmax group
+constexpr int TC_MAX_ILL = 32;       // ill-conditioned components the tensor-core assignment evaluates exactly for every point
 constexpr int64_t TC_YPOINTS = 1 << 19;   // points per launch of the tile kernel: capacity of the fp16 planes of Y in scratch
 constexpr size_t TC_YPLANE_BYTES = (size_t)TC_YPOINTS * 512;   // one plane: 256 fp16 values per point
 
@@ -35,6 +37,10 @@ struct TcBuffers {
     void* xl;   // exchange slots of the lower-bound pass
     unsigned char* y_hi;   // [TC_YPOINTS][256] fp16: high parts of Y = [s x | (s x)^2 + kap], k-step interleaved
     unsigned char* y_lo;   // the low parts
+    unsigned char* p_hi_rm;   // [Kpad][256] fp16: high parts of the scaled coefficients P / t_k, row-major, same column order as Y
+    unsigned char* p_lo_rm;   // the low parts
+    float* tkck;              // [Kpad] pairs (t_k, c_k); c_k = -inf for ill-conditioned components
+    int* ill_list;            // [Kpad] ascending indices of the ill-conditioned components (flags[2] of them)
 };
 
 bool tc_supports(int D, int K);
@@ -46,13 +52,22 @@ TcPlan tc_plan(int D, int K, int num_sms);
 size_t tc_scratch_bytes(int D, int K);
 cudaError_t tc_max_clusters(int D, int K, int* out);
 cudaError_t launch_prepare_tc(cudaStream_t s, int D, int K, const float* pi, const float* mu, const float* var,
-                              const TcBuffers& tb, float cond_limit, int* status);
+                              const TcBuffers& tb, float cond_limit, int* status, bool ill_list = false);
 // One pass over at most TC_YPOINTS points: X -> the two fp16 planes of Y in scratch (read by the tile kernel through TMA).
 cudaError_t launch_transform_tc(cudaStream_t s, const float* X, int64_t n, int D, const TcBuffers& tb);
 // n <= TC_YPOINTS points whose planes launch_transform_tc has written.
 // mu, w2, c2: the FP32 path's derived parameters (launch_prepare_fp32), used to recompute ill-conditioned logits exactly
 cudaError_t launch_em_tc(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu, const float* w2,
                          const float* c2, const TcBuffers& tb, int Q, int flush_tiles, int* status);
+// Tensor map of a plane [rows][256 halves] (Y or P): boxes of (one 128-byte atom row, box_rows rows, box_atoms atoms).
+cudaError_t tc_make_plane_map(CUtensorMap* tm, void* base, int64_t rows, int box_rows, int box_atoms);
+// Top-m assignment of n <= TC_YPOINTS points whose planes launch_transform_tc has written (tensor-core selection of
+// candidates + exact refinement).  rec: n * assign_tc_record_bytes(m) bytes of device scratch.  Needs launch_prepare_tc
+// with ill_list = true.  Both kernels return at once when tb.flags[3] != 0 (more than TC_MAX_ILL ill-conditioned
+// components): the caller then runs the FP32 kernels, gated the other way.
+size_t assign_tc_record_bytes(int m);
+cudaError_t launch_assign_tc(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu, const float* w2,
+                             const float* c2, const TcBuffers& tb, float* rec, int m, int32_t* idx, float* resp, int* status);
 cudaError_t launch_reduce_tc(cudaStream_t s, int D, int K, int Q, const TcBuffers& tb, double* Nk, double* S1,
                              double* S2, bool accumulate);
 

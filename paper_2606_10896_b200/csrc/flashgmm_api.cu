@@ -28,7 +28,7 @@ inline size_t align256(size_t b) { return (b + 255) & ~(size_t)255; }
 
 struct ScratchLayout {
     size_t w2, c2, c2d, partials, logZ2, llpart, result, stats, total;
-    size_t tc_phi, tc_plo, tc_tk, tc_ck, tc_sd, tc_kap, tc_illb, tc_flags, tc_xg, tc_xl, tc_partial, tc_llpart, tc_partial_bytes, tc_yhi, tc_ylo;
+    size_t tc_phi, tc_plo, tc_tk, tc_ck, tc_sd, tc_kap, tc_illb, tc_flags, tc_xg, tc_xl, tc_partial, tc_llpart, tc_partial_bytes, tc_yhi, tc_ylo, tc_phirm, tc_plorm, tc_tkck, tc_illlist;
     bool tc;
 };
 
@@ -47,7 +47,7 @@ ScratchLayout scratch_layout(int D, int K, bool planes) {
     L.result = take(sizeof(DevResult));
     L.stats = take(((size_t)K + 2 * KD) * 8);
     L.tc = tc_supports(D, K);
-    L.tc_phi = L.tc_plo = L.tc_tk = L.tc_ck = L.tc_sd = L.tc_kap = L.tc_illb = L.tc_flags = L.tc_xg = L.tc_xl = L.tc_partial = L.tc_llpart = L.tc_yhi = L.tc_ylo = 0;
+    L.tc_phi = L.tc_plo = L.tc_tk = L.tc_ck = L.tc_sd = L.tc_kap = L.tc_illb = L.tc_flags = L.tc_xg = L.tc_xl = L.tc_partial = L.tc_llpart = L.tc_yhi = L.tc_ylo = L.tc_phirm = L.tc_plorm = L.tc_tkck = L.tc_illlist = 0;
     L.tc_partial_bytes = 0;
     if (L.tc) {
         const TcPlan pl = tc_plan(D, K, 160);       // an upper bound on the number of clusters
@@ -64,6 +64,10 @@ ScratchLayout scratch_layout(int D, int K, bool planes) {
         L.tc_partial_bytes = (size_t)pl.Q * pl.Kpad * TC_PCOLS * 8;
         L.tc_partial = take(L.tc_partial_bytes);
         L.tc_llpart = take((size_t)pl.Q * 16);
+        L.tc_phirm = take((size_t)pl.Kpad * 512);
+        L.tc_plorm = take((size_t)pl.Kpad * 512);
+        L.tc_tkck = take((size_t)pl.Kpad * 8);
+        L.tc_illlist = take((size_t)pl.Kpad * 4);
     }
     if (L.tc && planes) {
         L.tc_yhi = take(TC_YPLANE_BYTES);
@@ -87,6 +91,8 @@ struct gmm_ctx {
     int capD = 0, capK = 0;
     void* pl_scratch = nullptr;      // posting-list builder: counters per (range of vectors, cluster)
     void* km_scratch = nullptr;      // k-means step: list offsets, per-segment float64 sums
+    void* at_scratch = nullptr;      // tensor-core assignment: candidate records of one piece of points
+    size_t at_scratch_bytes = 0;
     size_t km_scratch_bytes = 0;
     size_t pl_scratch_bytes = 0;
     bool capPlanes = false;    // the scratch layout in force includes the tensor path's planes of Y
@@ -136,6 +142,10 @@ struct gmm_ctx {
         b.llpart = reinterpret_cast<double*>(scratch + lay.tc_llpart);
         b.y_hi = scratch + lay.tc_yhi;
         b.y_lo = scratch + lay.tc_ylo;
+        b.p_hi_rm = scratch + lay.tc_phirm;
+        b.p_lo_rm = scratch + lay.tc_plorm;
+        b.tkck = reinterpret_cast<float*>(scratch + lay.tc_tkck);
+        b.ill_list = reinterpret_cast<int*>(scratch + lay.tc_illlist);
         return b;
     }
 };
@@ -399,6 +409,7 @@ int gmm_destroy(gmm_ctx* ctx) {
     if (ctx->hparams) cudaFree(ctx->hparams);
     if (ctx->pl_scratch) cudaFree(ctx->pl_scratch);
     if (ctx->km_scratch) cudaFree(ctx->km_scratch);
+    if (ctx->at_scratch) cudaFree(ctx->at_scratch);
     if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
     if (ctx->ev_created)
         for (int i = 0; i < EVENT_POOL; ++i) {
@@ -598,6 +609,10 @@ int gmm_em_step_host(gmm_ctx* ctx, const float* X_host, int64_t N, int D, int K,
     return read_result(ctx, 0, loglik);
 }
 
+namespace {
+int grow_buffer(gmm_ctx* ctx, void** buf, size_t* have, size_t need, const char* what);
+}
+
 int gmm_assign_topm(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const float* pi, const float* mu,
                     const float* var, int m, int32_t* idx, float* resp) {
     CHECK(check_shape(ctx, N, D, K));
@@ -612,11 +627,36 @@ int gmm_assign_topm(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const
     CHECK(ensure_scratch(ctx, D, K));
     CU(cudaMemsetAsync(&ctx->result()->status, 0, sizeof(int), ctx->stream));
     KL(launch_prepare_fp32(ctx->stream, D, K, pi, mu, var, ctx->w2(), ctx->c2(), ctx->c2d(), &ctx->result()->status));
+    // Tensor-core assignment where the E+M step would take the tensor path too.  Ill-conditioned components are evaluated
+    // exactly for every point; parameters with more than TC_MAX_ILL of them (a flag written on the device by the
+    // preparation kernels) go through the FP32 kernels instead: both sets of kernels are enqueued and each checks the
+    // flag, so the call stays asynchronous.
+    const bool tensor = ctx->capPlanes && ctx->lay.tc && ctx->path != GMM_PATH_FP32;
+    const int* run_fp32_if = nullptr;
+    if (tensor) {
+        const TcBuffers tb = ctx->tc();
+        const float limit = ctx->tc_cond_limit >= 0.f ? ctx->tc_cond_limit : 0.01f;
+        KL(launch_prepare_tc(ctx->stream, D, K, pi, mu, var, tb, limit, &ctx->result()->status, true));
+        ctx->launches += 2;
+        const int64_t piece = ctx->tc_piece;
+        const size_t need = (size_t)(N < piece ? N : piece) * assign_tc_record_bytes(m);
+        CHECK(grow_buffer(ctx, &ctx->at_scratch, &ctx->at_scratch_bytes, need, "the assignment records"));
+        for (int64_t off = 0; off < N; off += piece) {
+            const int64_t cnt = (N - off < piece) ? (N - off) : piece;
+            CHECK(prof_begin(ctx));
+            KL(launch_transform_tc(ctx->stream, X + off * D, cnt, D, tb));
+            KL(launch_assign_tc(ctx->stream, X + off * D, cnt, D, K, mu, ctx->w2(), ctx->c2(), tb,
+                                static_cast<float*>(ctx->at_scratch), m, idx + off * m, resp + off * m, &ctx->result()->status));
+            ctx->launches++;
+            CHECK(prof_end(ctx));
+        }
+        run_fp32_if = tb.flags + 3;
+    }
     for (int64_t off = 0; off < N; off += SUPER_TILE) {
         const int64_t cnt = (N - off < SUPER_TILE) ? (N - off) : SUPER_TILE;
-        KL(launch_topm_fp32(ctx->stream, X + off * D, cnt, D, K, mu, ctx->w2(), ctx->c2d(), m, idx + off * m, resp + off * m));
+        KL(launch_topm_fp32(ctx->stream, X + off * D, cnt, D, K, mu, ctx->w2(), ctx->c2d(), m, idx + off * m, resp + off * m, run_fp32_if));
     }
-    ctx->last_path = GMM_PATH_FP32;
+    ctx->last_path = tensor ? GMM_PATH_TENSOR : GMM_PATH_FP32;
     return GMM_OK;
 }
 

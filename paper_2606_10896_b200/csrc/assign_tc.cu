@@ -26,6 +26,9 @@
 
 #define TC_WAIT_LIMIT_NS 2000000000ull
 #include "tc_prims.cuh"
+#ifdef FLASHGMM_DEBUG
+#include <cstdlib>
+#endif
 
 namespace fg {
 
@@ -53,6 +56,9 @@ struct AssignParams {
     float* rec;                // [n][2][RECW] records (see assign_recw)
     int* status;
     const int* gate;           // the launch does nothing when gate[0] != 0 (too many ill-conditioned components: the FP32 kernels run instead)
+#ifdef FLASHGMM_DEBUG
+    int dbg;                   // what-if timing only (results are wrong): 1 no selection, 2 no softmax arithmetic, 4 no MMAs, 8 no B loads
+#endif
 };
 
 constexpr int assign_recw(int LIST) { return (2 + 2 * LIST + 3) & ~3; }      // words per record: m, s, LIST values, LIST indices
@@ -127,6 +133,9 @@ assign_tc_kernel(const AssignParams p, const __grid_constant__ CUtensorMap tm_yh
                         fence_before();
                         bar_arrive(BAR(AB_LEMPTY + grp));
                     }
+#ifdef FLASHGMM_DEBUG
+                    if (p.dbg & 2) continue;
+#endif
                     const int col0 = c * AT_COMPS + sub * 32;
                     const float4* tc4 = reinterpret_cast<const float4*>(p.tkck + col0);
                     float l[32];
@@ -150,6 +159,9 @@ assign_tc_kernel(const AssignParams p, const __grid_constant__ CUtensorMap tm_yh
                     }
                     s_run += acc0 + acc1;
                     // the LIST largest: most blocks hold nothing that beats any lane's current LIST-th value
+#ifdef FLASHGMM_DEBUG
+                    if (p.dbg & 1) continue;
+#endif
                     if (__any_sync(0xffffffffu, bmax > tv[LIST - 1])) {
 #pragma unroll
                         for (int j = 0; j < 32; ++j) {
@@ -218,9 +230,16 @@ assign_tc_kernel(const AssignParams p, const __grid_constant__ CUtensorMap tm_yh
                     if (use > 0 && !wait0(BAR(AB_BEMPTY + st), (uint32_t)((use - 1) & 1))) { ok = false; break; }
                     if (elect_one()) {
                         const uint32_t dst = smem_u32(smem + ASM_B + st * 2 * AT_ATOM);
+#ifdef FLASHGMM_DEBUG
+                        if (p.dbg & 8) bar_arrive(BAR(AB_BFULL + st));
+                        else {
+#endif
                         bar_expect_tx(BAR(AB_BFULL + st), 2 * AT_ATOM);
                         tma_load_3d(dst, &tm_phi, 0, c * AT_COMPS, a, BAR(AB_BFULL + st));
                         tma_load_3d(dst + AT_ATOM, &tm_plo, 0, c * AT_COMPS, a, BAR(AB_BFULL + st));
+#ifdef FLASHGMM_DEBUG
+                        }
+#endif
                     }
                     __syncwarp();
                     ++g;
@@ -270,6 +289,9 @@ assign_tc_kernel(const AssignParams p, const __grid_constant__ CUtensorMap tm_yh
                         const uint64_t ah = d_ahi + ((a * AT_ATOM) >> 4), al = d_alo + ((a * AT_ATOM) >> 4);
                         const uint64_t bh = d_b + ((st * 2 * AT_ATOM) >> 4), bl = bh + (AT_ATOM >> 4);
                         // the two small cross products first, then the leading one (as in the E-step of the tile kernel)
+#ifdef FLASHGMM_DEBUG
+                        if (!(p.dbg & 4)) {
+#endif
 #pragma unroll
                         for (int j = 0; j < 4; ++j)
                             if (j < kk) mma_ss(d, ah + ((j * 32) >> 4), bl + ((j * 32) >> 4), idesc, (a > 0 || j > 0) ? 1u : 0u);
@@ -279,6 +301,9 @@ assign_tc_kernel(const AssignParams p, const __grid_constant__ CUtensorMap tm_yh
 #pragma unroll
                         for (int j = 0; j < 4; ++j)
                             if (j < kk) mma_ss(d, ah + ((j * 32) >> 4), bh + ((j * 32) >> 4), idesc, 1u);
+#ifdef FLASHGMM_DEBUG
+                        }
+#endif
                         mma_commit(BAR(AB_BEMPTY + st));
                         if (c == NC - 1) mma_commit(BAR(AB_AEMPTY + a));
                         if (a == n_atoms - 1) mma_commit(BAR(AB_LFULL + b));
@@ -337,6 +362,41 @@ struct PointRow {
     }
 };
 
+// Warp-uniform list (every lane holds the same copy) of the GMM_MAX_TOPM largest exact values seen so far: descending,
+// equal values in ascending component order, whatever the order of insertion.
+struct ExactTop {
+    float v[GMM_MAX_TOPM];
+    int k[GMM_MAX_TOPM];
+    __device__ __forceinline__ void init() {
+#pragma unroll
+        for (int j = 0; j < GMM_MAX_TOPM; ++j) { v[j] = -CUDART_INF_F; k[j] = -1; }
+    }
+    __device__ __forceinline__ void insert(float e, int kk) {
+        constexpr int L = GMM_MAX_TOPM - 1;
+        if (!(k[L] < 0 || e > v[L] || (e == v[L] && kk < k[L]))) return;
+        v[L] = e; k[L] = kk;
+#pragma unroll
+        for (int j = L; j > 0; --j) {
+            if (k[j - 1] < 0 || v[j] > v[j - 1] || (v[j] == v[j - 1] && k[j] < k[j - 1])) {
+                const float fv = v[j]; v[j] = v[j - 1]; v[j - 1] = fv;
+                const int fk = k[j]; k[j] = k[j - 1]; k[j - 1] = fk;
+            }
+        }
+    }
+    __device__ __forceinline__ float value_at(int pos) const {
+        float r = -CUDART_INF_F;
+#pragma unroll
+        for (int j = 0; j < GMM_MAX_TOPM; ++j) if (j == pos) r = v[j];
+        return r;
+    }
+    __device__ __forceinline__ int index_at(int pos) const {
+        int r = -1;
+#pragma unroll
+        for (int j = 0; j < GMM_MAX_TOPM; ++j) if (j == pos) r = k[j];
+        return r;
+    }
+};
+
 template <int LIST>
 __global__ void __launch_bounds__(256)
 assign_refine_kernel(const float* __restrict__ rec, const float* __restrict__ X, int64_t n, int D, int K,
@@ -345,11 +405,22 @@ assign_refine_kernel(const float* __restrict__ rec, const float* __restrict__ X,
                      float* __restrict__ resp_out) {
     if (flags[3] != 0) return;
     constexpr int RECW = assign_recw(LIST);
-    constexpr int C = LIST - 1;                                  // candidates recomputed exactly
+    constexpr int C = LIST - 1;                                  // candidates that may be recomputed exactly
     const float e_launch = __int_as_float(flags[1]);             // error bound of the approximate logits from the parameters
-    const int n_ill = flags[2];                                  // ill-conditioned components (<= 32): always evaluated exactly
+    const int n_ill = flags[2];                                  // ill-conditioned components (<= 32): left out of the approximate pass
     const int lane = threadIdx.x & 31;
     const int ill_k = (lane < n_ill) ? __ldg(ill_list + lane) : -1;      // lane t keeps ill-conditioned component t
+    // first 8 dimensions of the ill-conditioned components (a cheap test, see below): [dimension][component]
+    __shared__ float ill_mu[8][32], ill_w[8][32], ill_c[32];
+    if (threadIdx.x < 32) {
+        const int k = (threadIdx.x < n_ill) ? __ldg(ill_list + threadIdx.x) : -1;
+        ill_c[threadIdx.x] = (k >= 0) ? __ldg(c2 + k) : -CUDART_INF_F;
+        for (int j = 0; j < 8; ++j) {
+            ill_mu[j][threadIdx.x] = (k >= 0 && j < D) ? __ldg(mu + (size_t)k * D + j) : 0.f;
+            ill_w[j][threadIdx.x] = (k >= 0 && j < D) ? __ldg(w2 + (size_t)k * D + j) : 0.f;
+        }
+    }
+    __syncthreads();
     const int64_t warp0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
     const float NEG = -CUDART_INF_F;
@@ -373,91 +444,89 @@ assign_refine_kernel(const float* __restrict__ rec, const float* __restrict__ X,
         }
         const int nvalid = __popc(__ballot_sync(0xffffffffu, ai >= 0));
         const int nc = nvalid < C ? nvalid : C;
+        auto approx_at = [&](int r) -> float {                    // approximate value of rank r, -inf when there is none
+            const unsigned b = __ballot_sync(0xffffffffu, ai >= 0 && rank == r);
+            const float v = __shfl_sync(0xffffffffu, av, b ? (__ffs(b) - 1) : 0);
+            return b ? v : NEG;
+        };
         PointRow pr;
         pr.load(X + row * D, D, lane);
-        // exact values of the candidates: lane r keeps candidate r (in the order of the approximate values)
+        ExactTop top;
+        top.init();
+
+        // Ill-conditioned components are evaluated exactly, unless their first 8 dimensions (kept in shared memory, lane t
+        // testing component t) already show that the component can neither reach the top m (its value stays below a lower
+        // bound of the m-th largest) nor weigh in the log-sum-exp (2^-40 of the largest term): a collapsed component is
+        // hopeless for every point but its own.
+        const float a_m = approx_at(m - 1);
+        const float skip_below = fminf(a_m - (e_launch + 1.f), fmaxf(m0, m1) - e_launch - 40.f);
+        float iv = NEG;
+        if (n_ill > 0) {
+            float part = 0.f;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const float xj = __shfl_sync(0xffffffffu, pr.x[0], j);          // dimension j (zero beyond D, where the weight is zero too)
+                const float diff = xj - ill_mu[j][lane];
+                part = fmaf(diff * diff, ill_w[j][lane], part);
+            }
+            // ill_c - part is an upper bound of the value: the other dimensions only lower it
+            unsigned alive_set = __ballot_sync(0xffffffffu, lane < n_ill && !(ill_c[lane] - part < skip_below));
+            while (alive_set) {
+                const int t = __ffs(alive_set) - 1;
+                alive_set &= alive_set - 1;
+                const int k = __shfl_sync(0xffffffffu, ill_k, t);
+                float mag;
+                const float e = __ldg(c2 + k) - pr.quad<false>(mu + (size_t)k * D, w2 + (size_t)k * D, D, lane, mag);
+                if (lane == t) iv = e;
+                if (e > NEG) top.insert(e, k);
+            }
+        }
+
+        // Candidates in the order of their approximate values, exactly; the walk stops as soon as the m-th largest exact
+        // value clears the next candidate's approximate value by more than the error bound (nothing further can enter)
+        // and that candidate no longer matters for the log-sum-exp.
+        // Error bound of an approximate logit: from the parameters (8 x the estimate, over the components of the
+        // approximate pass) plus from this point (8 x 2^-22 x the summed magnitude of the terms, largest so far).
         float ev = NEG, ea = NEG, tmax = 0.f;
-        int ek = -1;
+        bool stopped = false;
         for (int r = 0; r < nc; ++r) {
             const int src = __ffs(__ballot_sync(0xffffffffu, ai >= 0 && rank == r)) - 1;
             const int k = __shfl_sync(0xffffffffu, ai, src);
             const float a = __shfl_sync(0xffffffffu, av, src);
+            if (r >= m && top.index_at(m - 1) >= 0 && top.value_at(m - 1) > a + e_launch + 1.9073486e-06f * tmax &&
+                a < top.v[0] - 14.f) {                            // ... and it weighs less than 2^-14 of the largest term
+                stopped = true;
+                break;
+            }
             float mag;
-            const float q = pr.quad<true>(mu + (size_t)k * D, w2 + (size_t)k * D, D, lane, mag);
-            const float e = __ldg(c2 + k) - q;
+            const float e = __ldg(c2 + k) - pr.quad<true>(mu + (size_t)k * D, w2 + (size_t)k * D, D, lane, mag);
             tmax = fmaxf(tmax, mag);
-            if (lane == r) { ev = e; ea = a; ek = k; }
+            if (lane == r) { ev = e; ea = a; }
+            if (e > NEG) top.insert(e, k);
         }
-        // ... and of the ill-conditioned components, which the approximate pass left out (constant -inf there)
-        float iv = NEG;
-        for (int t = 0; t < n_ill; ++t) {
-            const int k = __shfl_sync(0xffffffffu, ill_k, t);
-            float mag;
-            const float q = pr.quad<false>(mu + (size_t)k * D, w2 + (size_t)k * D, D, lane, mag);
-            const float e = __ldg(c2 + k) - q;
-            if (lane == t) iv = e;
-        }
-        const int ik = (iv > NEG) ? ill_k : -1;                   // an ill-conditioned component of zero weight counts as absent here
-        float nxt = NEG;                                          // best approximate value outside the candidates
-        if (nvalid > C) {
-            const int src = __ffs(__ballot_sync(0xffffffffu, ai >= 0 && rank == C)) - 1;
-            nxt = __shfl_sync(0xffffffffu, av, src);
-        }
-        // order of all exactly known values (a lane holds up to two: a candidate and an ill-conditioned component)
-        int erank = 0, irank = 0;
-        const int span = (n_ill > 0) ? 32 : C;
-        for (int t = 0; t < span; ++t) {
-            const float ov = __shfl_sync(0xffffffffu, ev, t);
-            const int ok = __shfl_sync(0xffffffffu, ek, t);
-            if (ok >= 0) {
-                if (t != lane && (ek < 0 || ov > ev || (ov == ev && ok < ek))) ++erank;
-                if (ik < 0 || ov > iv || (ov == iv && ok < ik)) ++irank;
-            }
-            if (n_ill > 0) {
-                const float pv = __shfl_sync(0xffffffffu, iv, t);
-                const int pk = __shfl_sync(0xffffffffu, ik, t);
-                if (pk >= 0) {
-                    if (ek < 0 || pv > ev || (pv == ev && pk < ek)) ++erank;
-                    if (t != lane && (ik < 0 || pv > iv || (pv == iv && pk < ik))) ++irank;
-                }
-            }
-        }
-        const int nexact = __popc(__ballot_sync(0xffffffffu, ek >= 0)) + __popc(__ballot_sync(0xffffffffu, ik >= 0));
-        float e_m = NEG;                                          // m-th largest exact value
-        {
-            const unsigned b1 = __ballot_sync(0xffffffffu, ek >= 0 && erank == m - 1);
-            const unsigned b2 = __ballot_sync(0xffffffffu, ik >= 0 && irank == m - 1);
-            if (b1) e_m = __shfl_sync(0xffffffffu, ev, __ffs(b1) - 1);
-            else if (b2) e_m = __shfl_sync(0xffffffffu, iv, __ffs(b2) - 1);
-        }
-        // Error bound of an approximate logit: from the parameters (8 x the estimate, over the components that take part
-        // in the approximate pass) and from this point (8 x 2^-22 x the summed magnitude of the terms, largest over the
-        // candidates).
+        const float nxt = (nvalid > C) ? approx_at(C) : NEG;      // best approximate value outside the candidates
         const float ebound = e_launch + 1.9073486e-06f * tmax;
-        bool certain = nexact >= m && (nvalid <= C || e_m > nxt + ebound);
+        bool certain = top.index_at(m - 1) >= 0 && (stopped || nvalid <= C || top.value_at(m - 1) > nxt + ebound);
         float M = fmaxf(m0, m1), S = 0.f;
         if (certain) {
-            float emax = fmaxf(ev, iv);
+            M = fmaxf(M, top.v[0]);
+            // log-sum-exp: the approximate total with the evaluated candidates' approximate terms replaced by the exact
+            // ones, plus the ill-conditioned components.  The terms that stay approximate carry a relative error of a few
+            // 1e-4 each: the result is kept only if they make up less than a tenth of the total.
+            float ex = ((ev > NEG) ? fast_ex2(ev - M) : 0.f) + ((iv > NEG) ? fast_ex2(iv - M) : 0.f);
+            float ap = (ea > NEG) ? fast_ex2(ea - M) : 0.f;
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) emax = fmaxf(emax, __shfl_xor_sync(0xffffffffu, emax, o));
-            M = fmaxf(M, emax);
-            // log-sum-exp: the approximate total with the candidates' approximate terms replaced by the exact ones, plus
-            // the ill-conditioned components
-            float corr = (ek >= 0) ? (fast_ex2(ev - M) - fast_ex2(ea - M)) : 0.f;
-            if (ik >= 0) corr += fast_ex2(iv - M);
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) corr += __shfl_xor_sync(0xffffffffu, corr, o);
-            S = s0 * fast_ex2(m0 - M) + s1 * fast_ex2(m1 - M) + corr;
-            if (!(S > 0.f) || !(S < CUDART_INF_F)) certain = false;
+            for (int o = 16; o > 0; o >>= 1) {
+                ex += __shfl_xor_sync(0xffffffffu, ex, o);
+                ap += __shfl_xor_sync(0xffffffffu, ap, o);
+            }
+            S = (s0 * fast_ex2(m0 - M) + s1 * fast_ex2(m1 - M) - ap) + ex;
+            if (!(S > 0.f) || !(S < CUDART_INF_F) || !(S - ex <= 0.1f * S)) certain = false;
         }
         if (certain) {
-            if (ek >= 0 && erank < m) {
-                idx_out[row * m + erank] = ek;
-                resp_out[row * m + erank] = __fdividef(fast_ex2(ev - M), S);
-            }
-            if (ik >= 0 && irank < m) {
-                idx_out[row * m + irank] = ik;
-                resp_out[row * m + irank] = __fdividef(fast_ex2(iv - M), S);
+            if (lane < m) {
+                idx_out[row * m + lane] = top.index_at(lane);
+                resp_out[row * m + lane] = __fdividef(fast_ex2(top.value_at(lane) - M), S);
             }
             continue;
         }
@@ -505,6 +574,9 @@ cudaError_t launch_assign_t(cudaStream_t s, const float* X, int64_t n, int D, in
     p.n = n; p.n_chunks = pl.CL; p.n_ks = pl.n_ks;
     p.tkck = reinterpret_cast<const float2*>(tb.tkck);
     p.rec = rec; p.status = status; p.gate = tb.flags + 3;
+#ifdef FLASHGMM_DEBUG
+    p.dbg = std::getenv("GMM_AT_DBG") ? std::atoi(std::getenv("GMM_AT_DBG")) : 0;
+#endif
     const int64_t rows_padded = (n + TC_BN - 1) / TC_BN * TC_BN;       // what launch_transform_tc wrote
     CUtensorMap tm_yhi, tm_ylo, tm_phi, tm_plo;
     cudaError_t e = tc_make_plane_map(&tm_yhi, tb.y_hi, rows_padded, AT_POINTS, 1);
@@ -535,13 +607,16 @@ cudaError_t launch_assign_t(cudaStream_t s, const float* X, int64_t n, int D, in
 
 }  // namespace
 
-size_t assign_tc_record_bytes(int m) { return (size_t)2 * (m <= 4 ? assign_recw(8) : assign_recw(12)) * sizeof(float); }
+// LIST = 6 (m <= 4) or 10: the m wanted, at least one spare candidate, and the best value left outside (for the certainty
+// test).  Small m keeps 5 candidates too: the responsibilities are only as accurate as the share of the log-sum-exp that
+// the exactly evaluated components hold.
+size_t assign_tc_record_bytes(int m) { return (size_t)2 * assign_recw(m <= 4 ? 6 : 10) * sizeof(float); }
 
 cudaError_t launch_assign_tc(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu, const float* w2,
                              const float* c2, const TcBuffers& tb, float* rec, int m, int32_t* idx, float* resp, int* status) {
     if (n < 1 || n > TC_YPOINTS || m < 1 || m > GMM_MAX_TOPM) return cudaErrorInvalidValue;
-    if (m <= 4) return launch_assign_t<8>(s, X, n, D, K, mu, w2, c2, tb, rec, m, idx, resp, status);
-    return launch_assign_t<12>(s, X, n, D, K, mu, w2, c2, tb, rec, m, idx, resp, status);
+    if (m <= 4) return launch_assign_t<6>(s, X, n, D, K, mu, w2, c2, tb, rec, m, idx, resp, status);
+    return launch_assign_t<10>(s, X, n, D, K, mu, w2, c2, tb, rec, m, idx, resp, status);
 }
 
 }  // namespace fg

@@ -361,6 +361,80 @@ def test_topm_against_oracle(fg, ctx, cfg, n, m):
     assert_topm_matches(idx_g.cpu().numpy(), resp_g.cpu().numpy(), idx_r, resp_r, next_r, what=f"cfg {cfg} m {m}")
 
 
+def _random_mixture(rng, N, D, K, spread=2.0):
+    X = (rng.normal(size=(N, D)) * spread).astype(np.float32)
+    mu = (X[rng.choice(N, K, replace=K > N)] + 0.1 * rng.normal(size=(K, D))).astype(np.float32)
+    var = rng.uniform(0.5, 2.0, size=(K, D)).astype(np.float32)
+    pi = rng.dirichlet(np.ones(K)).astype(np.float32)
+    return X, pi, mu, var
+
+
+def _topm_tensor_vs_oracle(fg, ctx, X, pi, mu, var, m, what, expect_path=None):
+    ctx.gmm_set_path(fg.GMM_PATH_TENSOR)
+    idx_r, resp_r, next_r = orc.topm(X, pi, mu, var, m)
+    idx_g, resp_g = ctx.gmm_assign_topm(_t(X), _t(pi), _t(mu), _t(var), m)
+    torch.cuda.synchronize()
+    assert ctx.gmm_last_path() == (expect_path or fg.GMM_PATH_TENSOR)
+    assert_topm_matches(idx_g.cpu().numpy(), resp_g.cpu().numpy(), idx_r, resp_r, next_r, what=what)
+
+
+@pytest.mark.parametrize("N,D,K,m", [(1500, 128, 1024, 4), (777, 30, 100, 2), (2000, 100, 200, 8), (300, 9, 1000, 1),
+                                     (4097, 64, 640, 3), (129, 128, 64, 4), (1000, 128, 1024, 1)])
+def test_topm_tensor_path_against_oracle(fg, ctx, N, D, K, m):
+    """Tensor-core selection + exact refinement (Sections 4.2-4.3): several tiles of 128 points with a ragged tail, odd
+    numbers of 128-component chunks, dimensions that do not fill the 64-column atoms."""
+    X, pi, mu, var = _random_mixture(np.random.default_rng(N + D + K), N, D, K)
+    _topm_tensor_vs_oracle(fg, ctx, X, pi, mu, var, m, f"tensor top-m N={N} D={D} K={K} m={m}")
+
+
+def test_topm_tensor_path_after_em_iterations(fg, ctx):
+    spec = synth.CONFIGS[2].with_n(3000)
+    X = synth.sample_host(spec)
+    pi0, mu0, var0 = synth.init_params(X, spec)
+    for iters in (0, 3):            # broad posteriors at the initial parameters, sharp ones (and collapsed components) later
+        fit = orc.fit(X, pi0, mu0, var0, iters, var_floor=spec.var_floor) if iters else {"pi": pi0, "mu": mu0, "var": var0}
+        p32, m32, v32 = (np.asarray(fit[k], np.float32) for k in ("pi", "mu", "var"))
+        _topm_tensor_vs_oracle(fg, ctx, X, p32, m32, v32, 4, f"config 2 after {iters} iterations")
+
+
+def test_topm_tensor_path_degenerate_parameters(fg, ctx):
+    rng = np.random.default_rng(11)
+    N, D, K = 3000, 128, 256
+    X = rng.normal(size=(N, D)).astype(np.float32)
+    mu = X[:K].copy()
+    pi = np.full(K, 1 / K, np.float32)
+    var = np.ones((K, D), np.float32)
+    # a few components collapsed onto their point at the variance floor: evaluated exactly for every point
+    v = var.copy(); v[:5] = 1e-6
+    _topm_tensor_vs_oracle(fg, ctx, X, pi, mu, v, 4, "5 collapsed components")
+    # more of them than the tensor-core kernels take: the FP32 kernels run (decided on the device)
+    v = var.copy(); v[:40] = 1e-6
+    _topm_tensor_vs_oracle(fg, ctx, X, pi, mu, v, 4, "40 collapsed components")
+    # zero weights; exactly equal components (ties go to the smaller index); posteriors spread over hundreds of components
+    p2 = pi.copy(); p2[::2] = 0; p2 /= p2.sum()
+    _topm_tensor_vs_oracle(fg, ctx, X, p2, mu, var, 4, "zero weights")
+    m2 = mu.copy(); m2[10:20] = m2[10]
+    _topm_tensor_vs_oracle(fg, ctx, X, pi, m2, var, 8, "identical components")
+    _topm_tensor_vs_oracle(fg, ctx, X, pi, (mu * 0.01).astype(np.float32), var * 100, 4, "diffuse posteriors")
+    # all components identical: every point ties K ways
+    Xz = np.zeros((200, D), np.float32)
+    idx, resp = ctx.gmm_assign_topm(_t(Xz), _t(pi), _t(np.zeros((K, D))), _t(var), 3)
+    torch.cuda.synchronize()
+    assert np.array_equal(idx.cpu().numpy(), np.tile([0, 1, 2], (200, 1)))
+    np.testing.assert_allclose(resp.cpu().numpy(), 1 / K, rtol=1e-5)
+
+
+def test_topm_tensor_path_over_several_pieces(fg, ctx, monkeypatch):
+    """Pieces of 1024 points (instead of 2^19): the candidate records and the planes of Y are reused piece after piece."""
+    monkeypatch.setenv("GMM_TC_PIECE", "1024")
+    c2 = fg.Context(0)
+    try:
+        X, pi, mu, var = _random_mixture(np.random.default_rng(5), 2500, 64, 256)
+        _topm_tensor_vs_oracle(fg, c2, X, pi, mu, var, 2, "three pieces")
+    finally:
+        c2.close()
+
+
 def test_topm_exact_ties_go_to_the_smaller_index(fg, ctx):
     X = _t(np.zeros((70, 4), np.float32))
     K = 6

@@ -362,17 +362,25 @@ struct PointRow {
     }
 };
 
-// Warp-uniform list (every lane holds the same copy) of the GMM_MAX_TOPM largest exact values seen so far: descending,
-// equal values in ascending component order, whatever the order of insertion.
+#ifdef FLASHGMM_DEBUG
+__device__ unsigned long long g_refine_counts[4];     // sharp points, exact candidate evaluations, exact ill evaluations, full scans
+#define RCOUNT(i, v) do { if (lane == 0) atomicAdd(&g_refine_counts[i], (unsigned long long)(v)); } while (0)
+#else
+#define RCOUNT(i, v)
+#endif
+
+// Warp-uniform list (every lane holds the same copy) of the MAXM largest exact values seen so far: descending, equal
+// values in ascending component order, whatever the order of insertion.
+template <int MAXM>
 struct ExactTop {
-    float v[GMM_MAX_TOPM];
-    int k[GMM_MAX_TOPM];
+    float v[MAXM];
+    int k[MAXM];
     __device__ __forceinline__ void init() {
 #pragma unroll
-        for (int j = 0; j < GMM_MAX_TOPM; ++j) { v[j] = -CUDART_INF_F; k[j] = -1; }
+        for (int j = 0; j < MAXM; ++j) { v[j] = -CUDART_INF_F; k[j] = -1; }
     }
     __device__ __forceinline__ void insert(float e, int kk) {
-        constexpr int L = GMM_MAX_TOPM - 1;
+        constexpr int L = MAXM - 1;
         if (!(k[L] < 0 || e > v[L] || (e == v[L] && kk < k[L]))) return;
         v[L] = e; k[L] = kk;
 #pragma unroll
@@ -386,182 +394,315 @@ struct ExactTop {
     __device__ __forceinline__ float value_at(int pos) const {
         float r = -CUDART_INF_F;
 #pragma unroll
-        for (int j = 0; j < GMM_MAX_TOPM; ++j) if (j == pos) r = v[j];
+        for (int j = 0; j < MAXM; ++j) if (j == pos) r = v[j];
         return r;
     }
     __device__ __forceinline__ int index_at(int pos) const {
         int r = -1;
 #pragma unroll
-        for (int j = 0; j < GMM_MAX_TOPM; ++j) if (j == pos) r = k[j];
+        for (int j = 0; j < MAXM; ++j) if (j == pos) r = k[j];
         return r;
     }
 };
 
+// Per-thread sorted list of approximate values (descending, equal values in ascending component order).
 template <int LIST>
+struct ApproxList {
+    float a[LIST];
+    int i[LIST];
+    __device__ __forceinline__ void insert(float val, int id) {
+        constexpr int L = LIST - 1;
+        if (!(i[L] < 0 || val > a[L] || (val == a[L] && id < i[L]))) return;
+        a[L] = val; i[L] = id;
+#pragma unroll
+        for (int j = L; j > 0; --j) {
+            if (i[j - 1] < 0 || a[j] > a[j - 1] || (a[j] == a[j - 1] && i[j] < i[j - 1])) {
+                const float fv = a[j]; a[j] = a[j - 1]; a[j - 1] = fv;
+                const int fi = i[j]; i[j] = i[j - 1]; i[j - 1] = fi;
+            }
+        }
+    }
+};
+
+struct RefineArgs {
+    const float* X; int64_t n; int D, K;
+    const float* mu; const float* w2; const float* c2;
+    int m; int32_t* idx_out; float* resp_out;
+    float e_launch; int n_ill;
+};
+
+// One point, the whole warp: exact evaluation of what matters (see assign_refine_kernel).  Lane q < LIST holds the q-th
+// best approximate value sv and its component si of the point (-inf / -1 where there is none).
+template <int LIST, int MAXM>
+__device__ __forceinline__ void refine_point(const RefineArgs& g, const TcIllCache& ill, int64_t row, int lane, float sv, int si,
+                                             float m0, float s0, float m1, float s1) {
+    constexpr int C = LIST - 1;                                  // candidates that may be recomputed exactly
+    const float NEG = -CUDART_INF_F;
+    const int m = g.m, D = g.D;
+    const float e_launch = g.e_launch;
+    const int nvalid = __popc(__ballot_sync(0xffffffffu, si >= 0));
+    const int nc = nvalid < C ? nvalid : C;
+    // A component matters when its responsibility may exceed 2^-24 (6e-8): those are evaluated exactly.  Among the rest,
+    // order and values are those of the approximate pass (differences far below the 1e-6 tie width of the assignment).
+    const float a0 = __shfl_sync(0xffffffffu, sv, 0);
+    const float matter = a0 - e_launch - 25.f;
+    const int p = __popc(__ballot_sync(0xffffffffu, lane < nc && sv >= matter));      // a prefix: the values descend
+    PointRow pr;
+    pr.load(g.X + row * D, D, lane);
+    ExactTop<MAXM> top;
+    top.init();
+    int n_exact = 0;                                              // exact values inserted into `top`
+
+    // Ill-conditioned components are evaluated exactly, unless their 8 dimensions of largest weight (kept in shared
+    // memory, one component per lane) already show that the component can neither reach the top m (its value stays below
+    // a lower bound of the m-th largest) nor weigh in the log-sum-exp (2^-40 of the largest term): a component that has
+    // collapsed in some dimensions is hopeless for every point but its own.  Their terms of the log-sum-exp are summed
+    // on line: (Mi, Si).
+    float Mi = NEG, Si = 0.f;
+    if (g.n_ill > 0) {
+        const float a_m = __shfl_sync(0xffffffffu, sv, m - 1);
+        const float skip_below = fminf(a_m - (e_launch + 1.f), fmaxf(m0, m1) - e_launch - 40.f);
+        const float* xr = g.X + row * D;
+        for (int base = 0; base < g.n_ill; base += 32) {
+            const int t = base + lane;
+            float part = 0.f, cc = NEG;
+            if (t < g.n_ill) {
+                cc = ill.c[t];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const float diff = __ldg(xr + ill.dim[j][t]) - ill.mu[j][t];          // (the row sits in L1 by now)
+                    part = fmaf(diff * diff, ill.w[j][t], part);
+                }
+            }
+            // cc - part is an upper bound of the value: the other dimensions only lower it
+            unsigned alive_set = __ballot_sync(0xffffffffu, t < g.n_ill && !(cc - part < skip_below));
+            while (alive_set) {
+                const int k = ill.k[base + __ffs(alive_set) - 1];
+                alive_set &= alive_set - 1;
+                float mag;
+                const float e = __ldg(g.c2 + k) - pr.quad<false>(g.mu + (size_t)k * D, g.w2 + (size_t)k * D, D, lane, mag);
+                RCOUNT(2, 1);
+                if (e > NEG) {
+                    top.insert(e, k);
+                    ++n_exact;
+                    if (e > Mi) { Si = Si * fast_ex2(Mi - e) + 1.f; Mi = e; }
+                    else Si += fast_ex2(e - Mi);
+                }
+            }
+        }
+    }
+
+    // Candidates that matter, in the order of their approximate values, exactly.  A point with a single component that
+    // matters needs none: its responsibility is 1 - (what the approximate pass summed for the others).  The walk also
+    // stops at a candidate that can neither enter the top m (the m-th largest exact value clears its approximate value by
+    // more than the error bound) nor weigh in the log-sum-exp (2^-14 of the largest term).
+    // Error bound of an approximate logit: from the parameters (8 x the estimate, over the components of the approximate
+    // pass) plus from this point (8 x 2^-22 x the summed magnitude of the terms, largest so far).
+    float ev = NEG, ea = NEG, tmax = 0.f;
+    int evaluated = 0;
+    bool stopped = false;
+    if (p >= 2 || (p == 1 && n_exact > 0)) {
+        for (int r = 0; r < p; ++r) {
+            const float a = __shfl_sync(0xffffffffu, sv, r);
+            const int k = __shfl_sync(0xffffffffu, si, r);
+            if (r >= m && top.index_at(m - 1) >= 0 && top.value_at(m - 1) > a + e_launch + 1.9073486e-06f * tmax &&
+                a < top.v[0] - 14.f) {
+                stopped = true;
+                break;
+            }
+            float mag;
+            const float e = __ldg(g.c2 + k) - pr.quad<true>(g.mu + (size_t)k * D, g.w2 + (size_t)k * D, D, lane, mag);
+            RCOUNT(1, 1);
+            tmax = fmaxf(tmax, mag);
+            if (lane == r) { ev = e; ea = a; }
+            ++evaluated;
+            if (e > NEG) { top.insert(e, k); ++n_exact; }
+        }
+    }
+    const int n_top = n_exact < MAXM ? n_exact : MAXM;            // what the list holds
+    const float ebound = e_launch + 1.9073486e-06f * tmax;
+    const float next_a = __shfl_sync(0xffffffffu, sv, evaluated);      // best approximate value among what was not evaluated (lane LIST - 1 at most)
+    // The first m come from the exact list, then from the unevaluated candidates in approximate order.
+    bool certain = n_top + (nvalid - evaluated) >= m && (n_top >= m || nvalid <= C || next_a < matter || evaluated == 0);
+    if (certain && n_top >= m)
+        certain = stopped || next_a == NEG || next_a < matter || top.value_at(m - 1) > next_a + ebound;
+    float M = fmaxf(m0, m1), S = 0.f;
+    if (certain) {
+        if (n_top > 0) M = fmaxf(M, top.v[0]);
+        // log-sum-exp: the approximate total with the evaluated candidates' approximate terms replaced by the exact ones,
+        // plus the ill-conditioned components.  The terms that stay approximate carry a relative error of a few 1e-4
+        // each: where components were evaluated, the result is kept only if the others make up less than a tenth of the
+        // total.
+        float ex = (ev > NEG) ? fast_ex2(ev - M) : 0.f;
+        float ap = (ea > NEG) ? fast_ex2(ea - M) : 0.f;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            ex += __shfl_xor_sync(0xffffffffu, ex, o);
+            ap += __shfl_xor_sync(0xffffffffu, ap, o);
+        }
+        if (Si > 0.f) ex += Si * fast_ex2(Mi - M);
+        S = (s0 * fast_ex2(m0 - M) + s1 * fast_ex2(m1 - M) - ap) + ex;
+        if (!(S > 0.f) || !(S < CUDART_INF_F)) certain = false;
+        else if (evaluated > 0 && !(S - ex <= 0.1f * S)) certain = false;
+    }
+    if (certain) {
+        // lane j writes output j: from the exact list, then from the unevaluated candidates
+        int q = evaluated + lane - n_top;
+        q = q < 0 ? 0 : (q > 31 ? 31 : q);
+        const float va = __shfl_sync(0xffffffffu, sv, q);
+        const int ka = __shfl_sync(0xffffffffu, si, q);
+        const bool from_top = lane < n_top;
+        const float v = from_top ? top.value_at(lane) : va;
+        const int k = from_top ? top.index_at(lane) : ka;
+        if (lane < m) {
+            g.idx_out[row * m + lane] = k;
+            g.resp_out[row * m + lane] = __fdividef(fast_ex2(v - M), S);
+        }
+        return;
+    }
+    RCOUNT(3, 1);
+    // ---- not certain (near ties, exact ties, too few finite candidates, broad posteriors): all K components exactly ----
+    float tv[GMM_MAX_TOPM];
+    int ti[GMM_MAX_TOPM];
+#pragma unroll
+    for (int j = 0; j < GMM_MAX_TOPM; ++j) { tv[j] = NEG; ti[j] = -1; }
+    float Mx = NEG, Sx = 0.f;
+    for (int k = 0; k < g.K; ++k) {
+        float mag;
+        const float q = pr.quad<false>(g.mu + (size_t)k * D, g.w2 + (size_t)k * D, D, lane, mag);
+        const float e = __ldg(g.c2 + k) - q;
+        if (e > Mx) { Sx = Sx * fast_ex2(Mx - e) + 1.f; Mx = e; }        // (Mx = -inf: Sx is 0, and 0 * 2^-inf = 0)
+        else if (e > NEG) Sx += fast_ex2(e - Mx);
+        // the GMM_MAX_TOPM largest (their first m are the answer): descending order, equal values keep the smaller index
+        // first, -inf values fill a list that is not full yet
+        if (ti[GMM_MAX_TOPM - 1] < 0 || e > tv[GMM_MAX_TOPM - 1]) {
+            tv[GMM_MAX_TOPM - 1] = e;
+            ti[GMM_MAX_TOPM - 1] = k;
+#pragma unroll
+            for (int j = GMM_MAX_TOPM - 1; j > 0; --j) {
+                if (ti[j] >= 0 && (ti[j - 1] < 0 || tv[j] > tv[j - 1])) {
+                    const float fv = tv[j]; tv[j] = tv[j - 1]; tv[j - 1] = fv;
+                    const int fi = ti[j]; ti[j] = ti[j - 1]; ti[j - 1] = fi;
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < GMM_MAX_TOPM; ++j) {
+        if (j < m && lane == 0) {
+            g.idx_out[row * m + j] = ti[j] >= 0 ? ti[j] : 0;
+            g.resp_out[row * m + j] = (ti[j] >= 0 && tv[j] > NEG && Sx > 0.f) ? __fdividef(fast_ex2(tv[j] - Mx), Sx) : 0.f;
+        }
+    }
+}
+
+// A warp takes 32 consecutive points.  First every lane looks at one point on its own: it merges the records of the two
+// warpgroups and, if only one component matters for the point (the second best approximate value lies 25 + the error
+// bound below the best, and no ill-conditioned component passes the 8-dimension test), writes the answer straight from
+// the approximate values: the best responsibility is 1 - (the rest), the others are below 6e-8.  The points that are
+// left are then taken one after the other by the whole warp (refine_point).
+template <int LIST, int MAXM>
 __global__ void __launch_bounds__(256)
 assign_refine_kernel(const float* __restrict__ rec, const float* __restrict__ X, int64_t n, int D, int K,
                      const float* __restrict__ mu, const float* __restrict__ w2, const float* __restrict__ c2,
-                     const int* __restrict__ flags, const int* __restrict__ ill_list, int m, int32_t* __restrict__ idx_out,
+                     const int* __restrict__ flags, const TcIllCache* __restrict__ ill_cache, int m, int32_t* __restrict__ idx_out,
                      float* __restrict__ resp_out) {
     if (flags[3] != 0) return;
     constexpr int RECW = assign_recw(LIST);
-    constexpr int C = LIST - 1;                                  // candidates that may be recomputed exactly
-    const float e_launch = __int_as_float(flags[1]);             // error bound of the approximate logits from the parameters
-    const int n_ill = flags[2];                                  // ill-conditioned components (<= 32): left out of the approximate pass
+    RefineArgs g;
+    g.X = X; g.n = n; g.D = D; g.K = K; g.mu = mu; g.w2 = w2; g.c2 = c2; g.m = m; g.idx_out = idx_out; g.resp_out = resp_out;
+    g.e_launch = __int_as_float(flags[1]);          // error bound of the approximate logits from the parameters
+    g.n_ill = flags[2];                             // ill-conditioned components (<= TC_MAX_ILL): left out of the approximate pass
     const int lane = threadIdx.x & 31;
-    const int ill_k = (lane < n_ill) ? __ldg(ill_list + lane) : -1;      // lane t keeps ill-conditioned component t
-    // first 8 dimensions of the ill-conditioned components (a cheap test, see below): [dimension][component]
-    __shared__ float ill_mu[8][32], ill_w[8][32], ill_c[32];
-    if (threadIdx.x < 32) {
-        const int k = (threadIdx.x < n_ill) ? __ldg(ill_list + threadIdx.x) : -1;
-        ill_c[threadIdx.x] = (k >= 0) ? __ldg(c2 + k) : -CUDART_INF_F;
-        for (int j = 0; j < 8; ++j) {
-            ill_mu[j][threadIdx.x] = (k >= 0 && j < D) ? __ldg(mu + (size_t)k * D + j) : 0.f;
-            ill_w[j][threadIdx.x] = (k >= 0 && j < D) ? __ldg(w2 + (size_t)k * D + j) : 0.f;
-        }
+    __shared__ TcIllCache ill;
+    if (g.n_ill > 0) {
+        const int* src = reinterpret_cast<const int*>(ill_cache);
+        int* dst = reinterpret_cast<int*>(&ill);
+        for (int i = threadIdx.x; i < (int)(sizeof(TcIllCache) / 4); i += blockDim.x) dst[i] = __ldg(src + i);
     }
     __syncthreads();
     const int64_t warp0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
     const float NEG = -CUDART_INF_F;
-    for (int64_t row = warp0; row < n; row += nwarps) {
-        const float* r0 = rec + (size_t)row * 2 * RECW;
-        float av = NEG;
-        int ai = -1;
-        if (lane < 2 * LIST) {
-            const int h = lane / LIST, j = lane - h * LIST;
-            av = __ldg(r0 + h * RECW + 2 + j);
-            ai = __float_as_int(__ldg(r0 + h * RECW + 2 + LIST + j));
-        }
-        const float m0 = __ldg(r0), s0 = __ldg(r0 + 1), m1 = __ldg(r0 + RECW), s1 = __ldg(r0 + RECW + 1);
-        // rank inside the union of the two lists: descending approximate value, ties to the smaller index
-        int rank = 0;
+    for (int64_t base = warp0 * 32; base < n; base += nwarps * 32) {
+        const int64_t row = base + lane;
+        const bool valid = row < n;
+        ApproxList<LIST> al;
+        float m0 = -1e30f, s0 = 0.f, m1 = -1e30f, s1 = 0.f;
 #pragma unroll
-        for (int t = 0; t < 2 * LIST; ++t) {
-            const float ov = __shfl_sync(0xffffffffu, av, t);
-            const int oi = __shfl_sync(0xffffffffu, ai, t);
-            if (t != lane && oi >= 0 && (ai < 0 || ov > av || (ov == av && oi < ai))) ++rank;
-        }
-        const int nvalid = __popc(__ballot_sync(0xffffffffu, ai >= 0));
-        const int nc = nvalid < C ? nvalid : C;
-        auto approx_at = [&](int r) -> float {                    // approximate value of rank r, -inf when there is none
-            const unsigned b = __ballot_sync(0xffffffffu, ai >= 0 && rank == r);
-            const float v = __shfl_sync(0xffffffffu, av, b ? (__ffs(b) - 1) : 0);
-            return b ? v : NEG;
-        };
-        PointRow pr;
-        pr.load(X + row * D, D, lane);
-        ExactTop top;
-        top.init();
-
-        // Ill-conditioned components are evaluated exactly, unless their first 8 dimensions (kept in shared memory, lane t
-        // testing component t) already show that the component can neither reach the top m (its value stays below a lower
-        // bound of the m-th largest) nor weigh in the log-sum-exp (2^-40 of the largest term): a collapsed component is
-        // hopeless for every point but its own.
-        const float a_m = approx_at(m - 1);
-        const float skip_below = fminf(a_m - (e_launch + 1.f), fmaxf(m0, m1) - e_launch - 40.f);
-        float iv = NEG;
-        if (n_ill > 0) {
-            float part = 0.f;
+        for (int j = 0; j < LIST; ++j) { al.a[j] = NEG; al.i[j] = -1; }
+        if (valid) {
+            const float4* r4 = reinterpret_cast<const float4*>(rec + (size_t)row * 2 * RECW);
+            float w[2 * RECW];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const float xj = __shfl_sync(0xffffffffu, pr.x[0], j);          // dimension j (zero beyond D, where the weight is zero too)
-                const float diff = xj - ill_mu[j][lane];
-                part = fmaf(diff * diff, ill_w[j][lane], part);
+            for (int j = 0; j < 2 * RECW / 4; ++j) {
+                const float4 q = __ldg(r4 + j);
+                w[4 * j] = q.x; w[4 * j + 1] = q.y; w[4 * j + 2] = q.z; w[4 * j + 3] = q.w;
             }
-            // ill_c - part is an upper bound of the value: the other dimensions only lower it
-            unsigned alive_set = __ballot_sync(0xffffffffu, lane < n_ill && !(ill_c[lane] - part < skip_below));
-            while (alive_set) {
-                const int t = __ffs(alive_set) - 1;
-                alive_set &= alive_set - 1;
-                const int k = __shfl_sync(0xffffffffu, ill_k, t);
-                float mag;
-                const float e = __ldg(c2 + k) - pr.quad<false>(mu + (size_t)k * D, w2 + (size_t)k * D, D, lane, mag);
-                if (lane == t) iv = e;
-                if (e > NEG) top.insert(e, k);
+            m0 = w[0]; s0 = w[1]; m1 = w[RECW]; s1 = w[RECW + 1];
+#pragma unroll
+            for (int j = 0; j < LIST; ++j) { al.a[j] = w[2 + j]; al.i[j] = __float_as_int(w[2 + LIST + j]); }      // sorted already
+#pragma unroll
+            for (int j = 0; j < LIST; ++j) {
+                const int id = __float_as_int(w[RECW + 2 + LIST + j]);
+                if (id >= 0) al.insert(w[RECW + 2 + j], id);
             }
         }
-
-        // Candidates in the order of their approximate values, exactly; the walk stops as soon as the m-th largest exact
-        // value clears the next candidate's approximate value by more than the error bound (nothing further can enter)
-        // and that candidate no longer matters for the log-sum-exp.
-        // Error bound of an approximate logit: from the parameters (8 x the estimate, over the components of the
-        // approximate pass) plus from this point (8 x 2^-22 x the summed magnitude of the terms, largest so far).
-        float ev = NEG, ea = NEG, tmax = 0.f;
-        bool stopped = false;
-        for (int r = 0; r < nc; ++r) {
-            const int src = __ffs(__ballot_sync(0xffffffffu, ai >= 0 && rank == r)) - 1;
-            const int k = __shfl_sync(0xffffffffu, ai, src);
-            const float a = __shfl_sync(0xffffffffu, av, src);
-            if (r >= m && top.index_at(m - 1) >= 0 && top.value_at(m - 1) > a + e_launch + 1.9073486e-06f * tmax &&
-                a < top.v[0] - 14.f) {                            // ... and it weighs less than 2^-14 of the largest term
-                stopped = true;
-                break;
-            }
-            float mag;
-            const float e = __ldg(c2 + k) - pr.quad<true>(mu + (size_t)k * D, w2 + (size_t)k * D, D, lane, mag);
-            tmax = fmaxf(tmax, mag);
-            if (lane == r) { ev = e; ea = a; }
-            if (e > NEG) top.insert(e, k);
-        }
-        const float nxt = (nvalid > C) ? approx_at(C) : NEG;      // best approximate value outside the candidates
-        const float ebound = e_launch + 1.9073486e-06f * tmax;
-        bool certain = top.index_at(m - 1) >= 0 && (stopped || nvalid <= C || top.value_at(m - 1) > nxt + ebound);
-        float M = fmaxf(m0, m1), S = 0.f;
-        if (certain) {
-            M = fmaxf(M, top.v[0]);
-            // log-sum-exp: the approximate total with the evaluated candidates' approximate terms replaced by the exact
-            // ones, plus the ill-conditioned components.  The terms that stay approximate carry a relative error of a few
-            // 1e-4 each: the result is kept only if they make up less than a tenth of the total.
-            float ex = ((ev > NEG) ? fast_ex2(ev - M) : 0.f) + ((iv > NEG) ? fast_ex2(iv - M) : 0.f);
-            float ap = (ea > NEG) ? fast_ex2(ea - M) : 0.f;
+        int nv = 0;
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                ex += __shfl_xor_sync(0xffffffffu, ex, o);
-                ap += __shfl_xor_sync(0xffffffffu, ap, o);
-            }
-            S = (s0 * fast_ex2(m0 - M) + s1 * fast_ex2(m1 - M) - ap) + ex;
-            if (!(S > 0.f) || !(S < CUDART_INF_F) || !(S - ex <= 0.1f * S)) certain = false;
-        }
-        if (certain) {
-            if (lane < m) {
-                idx_out[row * m + lane] = top.index_at(lane);
-                resp_out[row * m + lane] = __fdividef(fast_ex2(top.value_at(lane) - M), S);
-            }
-            continue;
-        }
-        // ---- not certain (near ties, exact ties, too few finite candidates): all K components exactly ----
-        float tv[GMM_MAX_TOPM];
-        int ti[GMM_MAX_TOPM];
+        for (int j = 0; j < LIST; ++j) nv += (al.i[j] >= 0) ? 1 : 0;
+        bool sharp = valid && nv >= m && al.a[1] < al.a[0] - g.e_launch - 25.f;
+        if (sharp && g.n_ill > 0) {
+            float a_m = NEG;
 #pragma unroll
-        for (int j = 0; j < GMM_MAX_TOPM; ++j) { tv[j] = NEG; ti[j] = -1; }
-        float Mx = NEG, Sx = 0.f;
-        for (int k = 0; k < K; ++k) {
-            float mag;
-            const float q = pr.quad<false>(mu + (size_t)k * D, w2 + (size_t)k * D, D, lane, mag);
-            const float e = __ldg(c2 + k) - q;
-            if (e > Mx) { Sx = Sx * fast_ex2(Mx - e) + 1.f; Mx = e; }        // (Mx = -inf: Sx is 0, and 0 * 2^-inf = 0)
-            else if (e > NEG) Sx += fast_ex2(e - Mx);
-            // the GMM_MAX_TOPM largest (their first m are the answer): descending order, equal values keep the smaller index
-            // first, -inf values fill a list that is not full yet
-            if (ti[GMM_MAX_TOPM - 1] < 0 || e > tv[GMM_MAX_TOPM - 1]) {
-                tv[GMM_MAX_TOPM - 1] = e;
-                ti[GMM_MAX_TOPM - 1] = k;
+            for (int j = 0; j < LIST; ++j) if (j == m - 1) a_m = al.a[j];
+            const float skip_below = fminf(a_m - (g.e_launch + 1.f), fmaxf(m0, m1) - g.e_launch - 40.f);
+            const float* xr = X + row * D;
+            for (int t = 0; t < g.n_ill && sharp; ++t) {
+                // upper bound of the component's value from its dimensions of largest weight, the largest first: most
+                // components are out after one
+                float ub = ill.c[t];
+                bool out = false;
 #pragma unroll
-                for (int j = GMM_MAX_TOPM - 1; j > 0; --j) {
-                    if (ti[j] >= 0 && (ti[j - 1] < 0 || tv[j] > tv[j - 1])) {
-                        const float fv = tv[j]; tv[j] = tv[j - 1]; tv[j - 1] = fv;
-                        const int fi = ti[j]; ti[j] = ti[j - 1]; ti[j - 1] = fi;
+                for (int j = 0; j < 8; ++j) {
+                    if (!out) {
+                        const float diff = __ldg(xr + ill.dim[j][t]) - ill.mu[j][t];
+                        ub -= diff * diff * ill.w[j][t];
+                        out = ub < skip_below;
                     }
                 }
+                if (!out) sharp = false;
             }
         }
+        if (sharp) {
+            const float M = fmaxf(m0, m1);
+            const float S = s0 * fast_ex2(m0 - M) + s1 * fast_ex2(m1 - M);
 #pragma unroll
-        for (int j = 0; j < GMM_MAX_TOPM; ++j) {
-            if (j < m && lane == 0) {
-                idx_out[row * m + j] = ti[j] >= 0 ? ti[j] : 0;
-                resp_out[row * m + j] = (ti[j] >= 0 && tv[j] > NEG && Sx > 0.f) ? __fdividef(fast_ex2(tv[j] - Mx), Sx) : 0.f;
+            for (int j = 0; j < LIST; ++j) {
+                if (j < m) {
+                    idx_out[row * m + j] = al.i[j];
+                    resp_out[row * m + j] = __fdividef(fast_ex2(al.a[j] - M), S);
+                }
             }
+#ifdef FLASHGMM_DEBUG
+            atomicAdd(&g_refine_counts[0], 1ull);
+#endif
+        }
+        unsigned todo = __ballot_sync(0xffffffffu, valid && !sharp);
+        while (todo) {
+            const int src = __ffs(todo) - 1;
+            todo &= todo - 1;
+            float sv = NEG;
+            int si = -1;
+#pragma unroll
+            for (int q = 0; q < LIST; ++q) {
+                const float v = __shfl_sync(0xffffffffu, al.a[q], src);
+                const int i = __shfl_sync(0xffffffffu, al.i[q], src);
+                if (lane == q) { sv = v; si = i; }
+            }
+            refine_point<LIST, MAXM>(g, ill, base + src, lane, sv, si, __shfl_sync(0xffffffffu, m0, src),
+                                     __shfl_sync(0xffffffffu, s0, src), __shfl_sync(0xffffffffu, m1, src),
+                                     __shfl_sync(0xffffffffu, s1, src));
         }
     }
 }
@@ -599,13 +740,23 @@ cudaError_t launch_assign_t(cudaStream_t s, const float* X, int64_t n, int D, in
     assign_tc_kernel<LIST><<<grid, AT_THREADS, ASM_BYTES, s>>>(p, tm_yhi, tm_ylo, tm_phi, tm_plo);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    const int64_t warps_wanted = n < (int64_t)sms * 64 ? n : (int64_t)sms * 64;      // 8 CTAs of 8 warps per SM
+    const int64_t batches = (n + 31) / 32;                                         // a warp takes 32 points at a time
+    const int64_t warps_wanted = batches < (int64_t)sms * 64 ? batches : (int64_t)sms * 64;
     const unsigned rgrid = (unsigned)((warps_wanted + 7) / 8);
-    assign_refine_kernel<LIST><<<rgrid, 256, 0, s>>>(rec, X, n, D, K, mu, w2, c2, tb.flags, tb.ill_list, m, idx, resp);
+    assign_refine_kernel<LIST, (LIST <= 6 ? 4 : GMM_MAX_TOPM)><<<rgrid, 256, 0, s>>>(rec, X, n, D, K, mu, w2, c2, tb.flags, tb.ill_cache, m, idx,
+                                                                               resp);
     return cudaGetLastError();
 }
 
 }  // namespace
+
+#ifdef FLASHGMM_DEBUG
+extern "C" void gmm_debug_refine_counts(unsigned long long* out) {
+    cudaMemcpyFromSymbol(out, g_refine_counts, sizeof(g_refine_counts));
+    unsigned long long z[4] = {0, 0, 0, 0};
+    cudaMemcpyToSymbol(g_refine_counts, z, sizeof(z));
+}
+#endif
 
 // LIST = 6 (m <= 4) or 10: the m wanted, at least one spare candidate, and the best value left outside (for the certainty
 // test).  Small m keeps 5 candidates too: the responsibilities are only as accurate as the share of the log-sum-exp that

@@ -1131,6 +1131,42 @@ __global__ void __launch_bounds__(1024) tc_ill_list_kernel(int Kpad, const float
     if (k == 0) { flags[2] = total; flags[3] = total > TC_MAX_ILL ? 1 : 0; }
 }
 
+// One thread per listed ill-conditioned component: its 8 dimensions of largest weight, in descending order of the weight.
+__global__ void __launch_bounds__(TC_MAX_ILL) tc_ill_cache_kernel(int D, const float* __restrict__ mu, const float* __restrict__ w2,
+                                                                  const float* __restrict__ c2, const int* __restrict__ ill_list,
+                                                                  const int* __restrict__ flags, TcIllCache* __restrict__ out) {
+    const int t = threadIdx.x;
+    const int n_ill = flags[2] < TC_MAX_ILL ? flags[2] : TC_MAX_ILL;
+    if (t >= n_ill) return;
+    const int k = ill_list[t];
+    float bw[8];
+    int bd[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) { bw[j] = -1.f; bd[j] = 0; }
+    for (int d = 0; d < D; ++d) {
+        const float w = w2[(size_t)k * D + d];
+        if (w > bw[7]) {
+            bw[7] = w; bd[7] = d;
+#pragma unroll
+            for (int j = 7; j > 0; --j) {
+                if (bw[j] > bw[j - 1]) {
+                    const float fw = bw[j]; bw[j] = bw[j - 1]; bw[j - 1] = fw;
+                    const int fd = bd[j]; bd[j] = bd[j - 1]; bd[j - 1] = fd;
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const bool have = bw[j] >= 0.f;                 // fewer than 8 dimensions: the slot weighs nothing
+        out->dim[j][t] = bd[j];
+        out->w[j][t] = have ? bw[j] : 0.f;
+        out->mu[j][t] = have ? mu[(size_t)k * D + bd[j]] : 0.f;
+    }
+    out->c[t] = c2[k];
+    out->k[t] = k;
+}
+
 // stats (+)= sum over Q cluster partials (float64, fixed order), undoing the responsibility scale, the per-dimension
 // data scale and the interleaved column order.
 __global__ void tc_reduce_kernel(int D, int K, int Kpad, int Q, const double* __restrict__ partial,
@@ -1209,7 +1245,7 @@ size_t tc_scratch_bytes(int D, int K) {
     b += (size_t)pl.CL * 128 * 128 * 4;                    // P_hi image
     b += (size_t)pl.CL * 65536;                            // P_lo image
     b += (size_t)pl.Kpad * 4 * 2 + 512;                    // t_k, c_k, s_d
-    b += (size_t)pl.Kpad * (512 * 2 + 8 + 4);              // row-major P planes, (t_k, c_k) pairs, list of ill-conditioned components
+    b += (size_t)pl.Kpad * (512 * 2 + 8 + 4) + sizeof(TcIllCache);      // row-major P planes, (t_k, c_k) pairs, ill-conditioned components
     b += (size_t)pl.Q * pl.Kpad * TC_PCOLS * 8;            // float64 partials
     b += (size_t)pl.Q * 16;
     b += 5 * (size_t)pl.Q * 4 * pl.CL * 64 * 16;           // exchange slots
@@ -1232,6 +1268,11 @@ cudaError_t launch_prepare_tc(cudaStream_t s, int D, int K, const float* pi, con
     e = cudaGetLastError();
     if (e != cudaSuccess || !ill_list) return e;
     tc_ill_list_kernel<<<1, 1024, 0, s>>>(pl.Kpad, tb.illb, tb.ill_list, tb.flags);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_ill_cache_tc(cudaStream_t s, int D, const float* mu, const float* w2, const float* c2, const TcBuffers& tb) {
+    tc_ill_cache_kernel<<<1, TC_MAX_ILL, 0, s>>>(D, mu, w2, c2, tb.ill_list, tb.flags, tb.ill_cache);
     return cudaGetLastError();
 }
 

@@ -11,9 +11,17 @@ constexpr int TC_BN = 64;            // points per tile
 constexpr int TC_FLUSH = 64;         // tiles between flushes of the TMEM accumulators into float64 partials (even)
 constexpr float TC_RSCALE = 4096.f;  // responsibilities are scaled by this power of two before the fp16 split
 constexpr int TC_PCOLS = 258;        // columns of a partial row: 256 statistics columns + N_k of each softmax group
-constexpr int TC_MAX_ILL = 32;       // ill-conditioned components the tensor-core assignment evaluates exactly for every point
+constexpr int TC_MAX_ILL = 256;       // ill-conditioned components the tensor-core assignment evaluates exactly for every point
 constexpr int64_t TC_YPOINTS = 1 << 19;   // points per launch of the tile kernel: capacity of the fp16 planes of Y in scratch
 constexpr size_t TC_YPLANE_BYTES = (size_t)TC_YPOINTS * 512;   // one plane: 256 fp16 values per point
+
+// What the assignment kernels keep of every ill-conditioned component for a cheap first test: its 8 dimensions of largest
+// weight (log2 e / (2 var), descending), the mean and the weight there, and its constant.  [dimension slot][component]
+struct TcIllCache {
+    float mu[8][TC_MAX_ILL], w[8][TC_MAX_ILL], c[TC_MAX_ILL];
+    int dim[8][TC_MAX_ILL];
+    int k[TC_MAX_ILL];
+};
 
 struct TcPlan {
     int CL;     // CTAs per group = ceil(K / 128)
@@ -41,6 +49,7 @@ struct TcBuffers {
     unsigned char* p_lo_rm;   // the low parts
     float* tkck;              // [Kpad] pairs (t_k, c_k); c_k = -inf for ill-conditioned components
     int* ill_list;            // [Kpad] ascending indices of the ill-conditioned components (flags[2] of them)
+    TcIllCache* ill_cache;    // filled by launch_ill_cache_tc
 };
 
 bool tc_supports(int D, int K);
@@ -59,6 +68,9 @@ cudaError_t launch_transform_tc(cudaStream_t s, const float* X, int64_t n, int D
 // mu, w2, c2: the FP32 path's derived parameters (launch_prepare_fp32), used to recompute ill-conditioned logits exactly
 cudaError_t launch_em_tc(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu, const float* w2,
                          const float* c2, const TcBuffers& tb, int Q, int flush_tiles, int* status);
+// After launch_prepare_tc(..., ill_list = true): fills tb.ill_cache for the first min(flags[2], TC_MAX_ILL) listed components.
+// w2, c2: the FP32 path's derived parameters (launch_prepare_fp32).
+cudaError_t launch_ill_cache_tc(cudaStream_t s, int D, const float* mu, const float* w2, const float* c2, const TcBuffers& tb);
 // Tensor map of a plane [rows][256 halves] (Y or P): boxes of (one 128-byte atom row, box_rows rows, box_atoms atoms).
 cudaError_t tc_make_plane_map(CUtensorMap* tm, void* base, int64_t rows, int box_rows, int box_atoms);
 // Top-m assignment of n <= TC_YPOINTS points whose planes launch_transform_tc has written (tensor-core selection of

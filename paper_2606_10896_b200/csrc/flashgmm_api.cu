@@ -28,7 +28,7 @@ inline size_t align256(size_t b) { return (b + 255) & ~(size_t)255; }
 
 struct ScratchLayout {
     size_t w2, c2, c2d, partials, logZ2, llpart, result, stats, total;
-    size_t tc_phi, tc_plo, tc_tk, tc_ck, tc_sd, tc_kap, tc_illb, tc_flags, tc_xg, tc_xl, tc_partial, tc_llpart, tc_partial_bytes, tc_yhi, tc_ylo, tc_phirm, tc_plorm, tc_tkck, tc_illlist;
+    size_t tc_phi, tc_plo, tc_tk, tc_ck, tc_sd, tc_kap, tc_illb, tc_flags, tc_xg, tc_xl, tc_partial, tc_llpart, tc_partial_bytes, tc_yhi, tc_ylo, tc_phirm, tc_plorm, tc_tkck, tc_illlist, tc_illcache;
     bool tc;
 };
 
@@ -47,7 +47,7 @@ ScratchLayout scratch_layout(int D, int K, bool planes) {
     L.result = take(sizeof(DevResult));
     L.stats = take(((size_t)K + 2 * KD) * 8);
     L.tc = tc_supports(D, K);
-    L.tc_phi = L.tc_plo = L.tc_tk = L.tc_ck = L.tc_sd = L.tc_kap = L.tc_illb = L.tc_flags = L.tc_xg = L.tc_xl = L.tc_partial = L.tc_llpart = L.tc_yhi = L.tc_ylo = L.tc_phirm = L.tc_plorm = L.tc_tkck = L.tc_illlist = 0;
+    L.tc_phi = L.tc_plo = L.tc_tk = L.tc_ck = L.tc_sd = L.tc_kap = L.tc_illb = L.tc_flags = L.tc_xg = L.tc_xl = L.tc_partial = L.tc_llpart = L.tc_yhi = L.tc_ylo = L.tc_phirm = L.tc_plorm = L.tc_tkck = L.tc_illlist = L.tc_illcache = 0;
     L.tc_partial_bytes = 0;
     if (L.tc) {
         const TcPlan pl = tc_plan(D, K, 160);       // an upper bound on the number of clusters
@@ -68,6 +68,7 @@ ScratchLayout scratch_layout(int D, int K, bool planes) {
         L.tc_plorm = take((size_t)pl.Kpad * 512);
         L.tc_tkck = take((size_t)pl.Kpad * 8);
         L.tc_illlist = take((size_t)pl.Kpad * 4);
+        L.tc_illcache = take(sizeof(TcIllCache));
     }
     if (L.tc && planes) {
         L.tc_yhi = take(TC_YPLANE_BYTES);
@@ -146,6 +147,7 @@ struct gmm_ctx {
         b.p_lo_rm = scratch + lay.tc_plorm;
         b.tkck = reinterpret_cast<float*>(scratch + lay.tc_tkck);
         b.ill_list = reinterpret_cast<int*>(scratch + lay.tc_illlist);
+        b.ill_cache = reinterpret_cast<TcIllCache*>(scratch + lay.tc_illcache);
         return b;
     }
 };
@@ -638,6 +640,7 @@ int gmm_assign_topm(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const
         const float limit = ctx->tc_cond_limit >= 0.f ? ctx->tc_cond_limit : 0.01f;
         KL(launch_prepare_tc(ctx->stream, D, K, pi, mu, var, tb, limit, &ctx->result()->status, true));
         ctx->launches += 2;
+        KL(launch_ill_cache_tc(ctx->stream, D, mu, ctx->w2(), ctx->c2(), tb));
         const int64_t piece = ctx->tc_piece;
         const size_t need = (size_t)(N < piece ? N : piece) * assign_tc_record_bytes(m);
         CHECK(grow_buffer(ctx, &ctx->at_scratch, &ctx->at_scratch_bytes, need, "the assignment records"));

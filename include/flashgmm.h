@@ -130,9 +130,11 @@ int gmm_fit(gmm_ctx* ctx, const float* X, int64_t N, int D, int K,
  * Where the tensor-core path applies (same rule as gmm_em_step) the logits of all components come from the tensor cores
  * as a selection pass and the best few per point are recomputed exactly in fp32, so indices and values are those of the
  * FP32 kernels; a point whose selection is not certain within the error bound of the selection pass is evaluated
- * against all K components exactly.  Parameters with more than 32 ill-conditioned components run on the FP32 kernels
- * (decided on the device; gmm_last_path then still reports the tensor path).  The first call allocates a buffer of
- * 48 or 80 bytes (m <= 4, m > 4) per point of one piece of at most 2^19 points, outside gmm_scratch_bytes. */
+ * against all K components exactly; components whose responsibility for a point is below 4.8e-7 keep the order and
+ * the values of the selection pass (inside the 1e-6 tie width).  Parameters with more than 256 ill-conditioned
+ * components run on the FP32 kernels (decided on the device; gmm_last_path then still reports the tensor path).  The
+ * first call allocates a buffer of 128 or 192 bytes (m <= 4, m > 4) per point of one piece of at most 2^19 points,
+ * outside gmm_scratch_bytes. */
 int gmm_assign_topm(gmm_ctx* ctx, const float* X, int64_t N, int D, int K,
                     const float* pi, const float* mu, const float* var, int m,
                     int32_t* idx, float* resp);

@@ -330,28 +330,59 @@ assign_tc_kernel(const AssignParams p, const __grid_constant__ CUtensorMap tm_yh
 }
 
 // ---------------------------------------------------------------------------------------------------------------
-// Exact log2 z of (point, component) pairs by direct differences in fp32, one warp per point: lane l holds the
-// dimensions l, l + 32, l + 64, l + 96 of the point.
+// Exact log2 z of (point, component) pairs by direct differences in fp32, one warp per point.  Lane l holds the
+// dimensions 4 l .. 4 l + 3 of the point (16-byte loads; D a multiple of 4 and 16-byte aligned rows), else the
+// dimensions l, l + 32, l + 64, l + 96.
 struct PointRow {
     float x[4];
+    bool vec;
     __device__ __forceinline__ void load(const float* __restrict__ xr, int D, int lane) {
+        vec = (D % 4 == 0) && ((reinterpret_cast<uintptr_t>(xr) & 15) == 0);
+        if (vec) {
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (4 * lane < D) v = __ldg(reinterpret_cast<const float4*>(xr) + lane);
+            x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
+        } else {
 #pragma unroll
-        for (int j = 0; j < 4; ++j) x[j] = (lane + 32 * j < D) ? __ldg(xr + lane + 32 * j) : 0.f;
+            for (int j = 0; j < 4; ++j) x[j] = (lane + 32 * j < D) ? __ldg(xr + lane + 32 * j) : 0.f;
+        }
     }
-    // sum_d w (x - mu)^2 and, with MAG, sum_d w (|x| + |mu|)^2 (the size of the terms the expanded form adds up)
+    // this lane's share of sum_d w (x - mu)^2 and, with MAG, of sum_d w (|x| + |mu|)^2 (the size of the terms the
+    // expanded form adds up); mr, wr: rows of a [K][D] array whose base is 16-byte aligned
     template <bool MAG>
-    __device__ __forceinline__ float quad(const float* __restrict__ mr, const float* __restrict__ wr, int D, int lane, float& mag) const {
+    __device__ __forceinline__ float partial(const float* __restrict__ mr, const float* __restrict__ wr, int D, int lane, float& mag) const {
         float q = 0.f, t = 0.f;
+        if (vec) {
+            if (4 * lane < D) {
+                const float4 m4 = __ldg(reinterpret_cast<const float4*>(mr) + lane);
+                const float4 w4 = __ldg(reinterpret_cast<const float4*>(wr) + lane);
+                const float mm[4] = {m4.x, m4.y, m4.z, m4.w}, ww[4] = {w4.x, w4.y, w4.z, w4.w};
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int d = lane + 32 * j;
-            if (d < D) {
-                const float mu = __ldg(mr + d), w = __ldg(wr + d);
-                const float diff = x[j] - mu;
-                q = fmaf(diff * diff, w, q);
-                if (MAG) { const float a = fabsf(x[j]) + fabsf(mu); t = fmaf(a * a, w, t); }
+                for (int j = 0; j < 4; ++j) {
+                    const float diff = x[j] - mm[j];
+                    q = fmaf(diff * diff, ww[j], q);
+                    if (MAG) { const float a = fabsf(x[j]) + fabsf(mm[j]); t = fmaf(a * a, ww[j], t); }
+                }
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int d = lane + 32 * j;
+                if (d < D) {
+                    const float mu = __ldg(mr + d), w = __ldg(wr + d);
+                    const float diff = x[j] - mu;
+                    q = fmaf(diff * diff, w, q);
+                    if (MAG) { const float a = fabsf(x[j]) + fabsf(mu); t = fmaf(a * a, w, t); }
+                }
             }
         }
+        mag = t;
+        return q;
+    }
+    template <bool MAG>
+    __device__ __forceinline__ float quad(const float* __restrict__ mr, const float* __restrict__ wr, int D, int lane, float& mag) const {
+        float t;
+        float q = partial<MAG>(mr, wr, D, lane, t);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
             q += __shfl_xor_sync(0xffffffffu, q, o);
@@ -442,10 +473,10 @@ __device__ __forceinline__ void refine_point(const RefineArgs& g, const TcIllCac
     const float e_launch = g.e_launch;
     const int nvalid = __popc(__ballot_sync(0xffffffffu, si >= 0));
     const int nc = nvalid < C ? nvalid : C;
-    // A component matters when its responsibility may exceed 2^-24 (6e-8): those are evaluated exactly.  Among the rest,
-    // order and values are those of the approximate pass (differences far below the 1e-6 tie width of the assignment).
+    // A component matters when its responsibility may exceed 2^-21 (4.8e-7): those are evaluated exactly.  Among the rest,
+    // order and values are those of the approximate pass (differences below the 1e-6 tie width of the assignment).
     const float a0 = __shfl_sync(0xffffffffu, sv, 0);
-    const float matter = a0 - e_launch - 25.f;
+    const float matter = a0 - e_launch - 21.f;
     const int p = __popc(__ballot_sync(0xffffffffu, lane < nc && sv >= matter));      // a prefix: the values descend
     PointRow pr;
     pr.load(g.X + row * D, D, lane);
@@ -492,32 +523,46 @@ __device__ __forceinline__ void refine_point(const RefineArgs& g, const TcIllCac
         }
     }
 
-    // Candidates that matter, in the order of their approximate values, exactly.  A point with a single component that
-    // matters needs none: its responsibility is 1 - (what the approximate pass summed for the others).  The walk also
-    // stops at a candidate that can neither enter the top m (the m-th largest exact value clears its approximate value by
-    // more than the error bound) nor weigh in the log-sum-exp (2^-14 of the largest term).
+    // Candidates that matter, exactly, all of them at once (their loads and reductions overlap).  A point with a single
+    // component that matters needs none: its responsibility is 1 - (what the approximate pass summed for the others).
     // Error bound of an approximate logit: from the parameters (8 x the estimate, over the components of the approximate
-    // pass) plus from this point (8 x 2^-22 x the summed magnitude of the terms, largest so far).
+    // pass) plus from this point (8 x 2^-22 x the summed magnitude of the terms of the best candidate, doubled for the
+    // others).
     float ev = NEG, ea = NEG, tmax = 0.f;
     int evaluated = 0;
-    bool stopped = false;
+    const bool stopped = false;
     if (p >= 2 || (p == 1 && n_exact > 0)) {
-        for (int r = 0; r < p; ++r) {
-            const float a = __shfl_sync(0xffffffffu, sv, r);
-            const int k = __shfl_sync(0xffffffffu, si, r);
-            if (r >= m && top.index_at(m - 1) >= 0 && top.value_at(m - 1) > a + e_launch + 1.9073486e-06f * tmax &&
-                a < top.v[0] - 14.f) {
-                stopped = true;
-                break;
+        float qv[C];
+        int kv[C];
+        float mag0 = 0.f;
+#pragma unroll
+        for (int r = 0; r < C; ++r) {
+            kv[r] = __shfl_sync(0xffffffffu, si, r);
+            qv[r] = 0.f;
+            if (r < p) {
+                float mg;
+                if (r == 0) { qv[r] = pr.partial<true>(g.mu + (size_t)kv[r] * D, g.w2 + (size_t)kv[r] * D, D, lane, mg); mag0 = mg; }
+                else qv[r] = pr.partial<false>(g.mu + (size_t)kv[r] * D, g.w2 + (size_t)kv[r] * D, D, lane, mg);
             }
-            float mag;
-            const float e = __ldg(g.c2 + k) - pr.quad<true>(g.mu + (size_t)k * D, g.w2 + (size_t)k * D, D, lane, mag);
-            RCOUNT(1, 1);
-            tmax = fmaxf(tmax, mag);
-            if (lane == r) { ev = e; ea = a; }
-            ++evaluated;
-            if (e > NEG) { top.insert(e, k); ++n_exact; }
         }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            mag0 += __shfl_xor_sync(0xffffffffu, mag0, o);
+#pragma unroll
+            for (int r = 0; r < C; ++r)
+                if (r < p) qv[r] += __shfl_xor_sync(0xffffffffu, qv[r], o);
+        }
+        tmax = 2.f * mag0;
+#pragma unroll
+        for (int r = 0; r < C; ++r) {
+            if (r < p) {
+                const float e = __ldg(g.c2 + kv[r]) - qv[r];
+                RCOUNT(1, 1);
+                if (lane == r) { ev = e; ea = sv; }
+                if (e > NEG) { top.insert(e, kv[r]); ++n_exact; }
+            }
+        }
+        evaluated = p;
     }
     const int n_top = n_exact < MAXM ? n_exact : MAXM;            // what the list holds
     const float ebound = e_launch + 1.9073486e-06f * tmax;
@@ -597,7 +642,7 @@ __device__ __forceinline__ void refine_point(const RefineArgs& g, const TcIllCac
 }
 
 // A warp takes 32 consecutive points.  First every lane looks at one point on its own: it merges the records of the two
-// warpgroups and, if only one component matters for the point (the second best approximate value lies 25 + the error
+// warpgroups and, if only one component matters for the point (the second best approximate value lies 21 + the error
 // bound below the best, and no ill-conditioned component passes the 8-dimension test), writes the answer straight from
 // the approximate values: the best responsibility is 1 - (the rest), the others are below 6e-8.  The points that are
 // left are then taken one after the other by the whole warp (refine_point).
@@ -651,7 +696,7 @@ assign_refine_kernel(const float* __restrict__ rec, const float* __restrict__ X,
         int nv = 0;
 #pragma unroll
         for (int j = 0; j < LIST; ++j) nv += (al.i[j] >= 0) ? 1 : 0;
-        bool sharp = valid && nv >= m && al.a[1] < al.a[0] - g.e_launch - 25.f;
+        bool sharp = valid && nv >= m && al.a[1] < al.a[0] - g.e_launch - 21.f;
         if (sharp && g.n_ill > 0) {
             float a_m = NEG;
 #pragma unroll

@@ -407,9 +407,13 @@ def test_topm_tensor_path_degenerate_parameters(fg, ctx):
     # a few components collapsed onto their point at the variance floor: evaluated exactly for every point
     v = var.copy(); v[:5] = 1e-6
     _topm_tensor_vs_oracle(fg, ctx, X, pi, mu, v, 4, "5 collapsed components")
-    # more of them than the tensor-core kernels take: the FP32 kernels run (decided on the device)
     v = var.copy(); v[:40] = 1e-6
-    _topm_tensor_vs_oracle(fg, ctx, X, pi, mu, v, 4, "40 collapsed components")
+    v[40:60, ::7] = 1e-4            # narrow in some dimensions only: the cheap test must look at those
+    _topm_tensor_vs_oracle(fg, ctx, X, pi, mu, v, 4, "60 ill-conditioned components")
+    # more of them than the tensor-core kernels take (256): the FP32 kernels run (decided on the device)
+    X5, pi5, mu5, var5 = _random_mixture(np.random.default_rng(12), 2000, 64, 512, spread=1.0)
+    var5[:300] = 1e-6
+    _topm_tensor_vs_oracle(fg, ctx, X5, pi5, mu5, var5, 2, "300 collapsed components")
     # zero weights; exactly equal components (ties go to the smaller index); posteriors spread over hundreds of components
     p2 = pi.copy(); p2[::2] = 0; p2 /= p2.sum()
     _topm_tensor_vs_oracle(fg, ctx, X, p2, mu, var, 4, "zero weights")

@@ -41,6 +41,8 @@ def parse():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--path", default="auto", choices=["auto", "fp32", "tensor"])
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--assign-m", type=int, default=0,
+                    help="also time gmm_assign_topm with this m on the same X (after the EM steps; reported as 'assign_topm')")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
 
@@ -268,6 +270,27 @@ def main():
         "ex2_per_s": N * K / (kern_ms_step * 1e-3),
     }
 
+    # ---- optional: the top-m assignment pass over the same X, under the parameters the EM steps left ----
+    assign = None
+    if args.assign_m > 0:
+        m = args.assign_m
+        idx = torch.empty((N, m), dtype=torch.int32, device=dev)
+        resp = torch.empty((N, m), dtype=torch.float32, device=dev)
+        ctx.gmm_assign_topm(X, pi, mu, var, m, out=(idx, resp))           # warm-up (allocates the record buffer)
+        torch.cuda.synchronize()
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = max(1, min(args.steps, 3))
+        a0.record()
+        for _ in range(reps):
+            ctx.gmm_assign_topm(X, pi, mu, var, m, out=(idx, resp))
+        a1.record()
+        torch.cuda.synchronize()
+        a_ms = a0.elapsed_time(a1) / reps
+        assign = {"m": m, "ms": a_ms, "points_per_s": N / (a_ms * 1e-3), "algorithmic_tflops": 4.0 * N * K * D / (a_ms * 1e-3) / 1e12,
+                  "path": "tensor" if ctx.gmm_last_path() == fg.GMM_PATH_TENSOR else "fp32",
+                  "mean_top1_resp": float(resp[:, 0].mean().item())}
+        del idx, resp
+
     # ---- end to end through the C ABI with HOST buffers (copies inside the timed region) ----
     e2e = None
     if not args.no_e2e:
@@ -339,7 +362,7 @@ def main():
             "point_component_dim_per_s": N_global * K * D / (ms_step * 1e-3),
             "algorithmic_tflops": 8.0 * N_global * K * D / (ms_step * 1e-3) / 1e12,
             "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": int(launches),
-            "clocks": clocks, "scratch_bytes": int(mem_extra),
+            "clocks": clocks, "scratch_bytes": int(mem_extra), "assign_topm": assign,
             "loglik_first_last": [trace[0], trace[-1]],
             "paper_context": {"A100_ms_per_iter_N1M": 3755.0 / 30, "A100_ms_per_iter_N100M": 74270.0 / 30},
         }

@@ -19,8 +19,9 @@
 //                      log-sum-exp by the difference between exact and approximate candidate terms, orders by the exact
 //                      values (ties to the smaller index) and writes the top m.  The selection is certain when the m-th
 //                      exact value clears the best non-candidate's approximate value by more than the error bound of the
-//                      approximation; otherwise (near ties, exact ties, fewer than m finite candidates) the warp
-//                      walks over all K components exactly.
+//                      approximation; otherwise (near ties, exact ties, fewer than m finite candidates, broad
+//                      posteriors) the row is put on a list, and the FP32 tile kernel evaluates the listed rows against
+//                      all K components afterwards.
 #include "internal.cuh"
 #include "em_tc.cuh"
 
@@ -460,6 +461,7 @@ struct RefineArgs {
     const float* mu; const float* w2; const float* c2;
     int m; int32_t* idx_out; float* resp_out;
     float e_launch; int n_ill;
+    int32_t* unc_rows; int* unc_count;      // rows left to the exact kernel, and their number
 };
 
 // One point, the whole warp: exact evaluation of what matters (see assign_refine_kernel).  Lane q < LIST holds the q-th
@@ -606,39 +608,10 @@ __device__ __forceinline__ void refine_point(const RefineArgs& g, const TcIllCac
         return;
     }
     RCOUNT(3, 1);
-    // ---- not certain (near ties, exact ties, too few finite candidates, broad posteriors): all K components exactly ----
-    float tv[GMM_MAX_TOPM];
-    int ti[GMM_MAX_TOPM];
-#pragma unroll
-    for (int j = 0; j < GMM_MAX_TOPM; ++j) { tv[j] = NEG; ti[j] = -1; }
-    float Mx = NEG, Sx = 0.f;
-    for (int k = 0; k < g.K; ++k) {
-        float mag;
-        const float q = pr.quad<false>(g.mu + (size_t)k * D, g.w2 + (size_t)k * D, D, lane, mag);
-        const float e = __ldg(g.c2 + k) - q;
-        if (e > Mx) { Sx = Sx * fast_ex2(Mx - e) + 1.f; Mx = e; }        // (Mx = -inf: Sx is 0, and 0 * 2^-inf = 0)
-        else if (e > NEG) Sx += fast_ex2(e - Mx);
-        // the GMM_MAX_TOPM largest (their first m are the answer): descending order, equal values keep the smaller index
-        // first, -inf values fill a list that is not full yet
-        if (ti[GMM_MAX_TOPM - 1] < 0 || e > tv[GMM_MAX_TOPM - 1]) {
-            tv[GMM_MAX_TOPM - 1] = e;
-            ti[GMM_MAX_TOPM - 1] = k;
-#pragma unroll
-            for (int j = GMM_MAX_TOPM - 1; j > 0; --j) {
-                if (ti[j] >= 0 && (ti[j - 1] < 0 || tv[j] > tv[j - 1])) {
-                    const float fv = tv[j]; tv[j] = tv[j - 1]; tv[j - 1] = fv;
-                    const int fi = ti[j]; ti[j] = ti[j - 1]; ti[j - 1] = fi;
-                }
-            }
-        }
-    }
-#pragma unroll
-    for (int j = 0; j < GMM_MAX_TOPM; ++j) {
-        if (j < m && lane == 0) {
-            g.idx_out[row * m + j] = ti[j] >= 0 ? ti[j] : 0;
-            g.resp_out[row * m + j] = (ti[j] >= 0 && tv[j] > NEG && Sx > 0.f) ? __fdividef(fast_ex2(tv[j] - Mx), Sx) : 0.f;
-        }
-    }
+    // Not certain (near ties, exact ties, too few finite candidates, broad posteriors): the point joins the list of rows
+    // that the FP32 tile kernel evaluates against all K components afterwards.  (The order of the list varies from run to
+    // run; the result of a row does not depend on it.)
+    if (lane == 0) g.unc_rows[atomicAdd(g.unc_count, 1)] = (int32_t)row;
 }
 
 // A warp takes 32 consecutive points.  First every lane looks at one point on its own: it merges the records of the two
@@ -651,10 +624,11 @@ __global__ void __launch_bounds__(256)
 assign_refine_kernel(const float* __restrict__ rec, const float* __restrict__ X, int64_t n, int D, int K,
                      const float* __restrict__ mu, const float* __restrict__ w2, const float* __restrict__ c2,
                      const int* __restrict__ flags, const TcIllCache* __restrict__ ill_cache, int m, int32_t* __restrict__ idx_out,
-                     float* __restrict__ resp_out) {
+                     float* __restrict__ resp_out, int32_t* __restrict__ unc_rows, int* __restrict__ unc_count) {
     if (flags[3] != 0) return;
     constexpr int RECW = assign_recw(LIST);
     RefineArgs g;
+    g.unc_rows = unc_rows; g.unc_count = unc_count;
     g.X = X; g.n = n; g.D = D; g.K = K; g.mu = mu; g.w2 = w2; g.c2 = c2; g.m = m; g.idx_out = idx_out; g.resp_out = resp_out;
     g.e_launch = __int_as_float(flags[1]);          // error bound of the approximate logits from the parameters
     g.n_ill = flags[2];                             // ill-conditioned components (<= TC_MAX_ILL): left out of the approximate pass
@@ -754,7 +728,8 @@ assign_refine_kernel(const float* __restrict__ rec, const float* __restrict__ X,
 
 template <int LIST>
 cudaError_t launch_assign_t(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu, const float* w2,
-                            const float* c2, const TcBuffers& tb, float* rec, int m, int32_t* idx, float* resp, int* status) {
+                            const float* c2, const TcBuffers& tb, float* rec, int32_t* unc_rows, int* unc_count, int m, int32_t* idx,
+                            float* resp, int* status) {
     const TcPlan pl = tc_plan(D, K, 148);
     AssignParams p;
     p.n = n; p.n_chunks = pl.CL; p.n_ks = pl.n_ks;
@@ -785,11 +760,13 @@ cudaError_t launch_assign_t(cudaStream_t s, const float* X, int64_t n, int D, in
     assign_tc_kernel<LIST><<<grid, AT_THREADS, ASM_BYTES, s>>>(p, tm_yhi, tm_ylo, tm_phi, tm_plo);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
+    e = cudaMemsetAsync(unc_count, 0, sizeof(int), s);
+    if (e != cudaSuccess) return e;
     const int64_t batches = (n + 31) / 32;                                         // a warp takes 32 points at a time
     const int64_t warps_wanted = batches < (int64_t)sms * 64 ? batches : (int64_t)sms * 64;
     const unsigned rgrid = (unsigned)((warps_wanted + 7) / 8);
     assign_refine_kernel<LIST, (LIST <= 6 ? 4 : GMM_MAX_TOPM)><<<rgrid, 256, 0, s>>>(rec, X, n, D, K, mu, w2, c2, tb.flags, tb.ill_cache, m, idx,
-                                                                               resp);
+                                                                               resp, unc_rows, unc_count);
     return cudaGetLastError();
 }
 
@@ -809,10 +786,11 @@ extern "C" void gmm_debug_refine_counts(unsigned long long* out) {
 size_t assign_tc_record_bytes(int m) { return (size_t)2 * assign_recw(m <= 4 ? 6 : 10) * sizeof(float); }
 
 cudaError_t launch_assign_tc(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu, const float* w2,
-                             const float* c2, const TcBuffers& tb, float* rec, int m, int32_t* idx, float* resp, int* status) {
+                             const float* c2, const TcBuffers& tb, float* rec, int32_t* unc_rows, int* unc_count, int m, int32_t* idx,
+                             float* resp, int* status) {
     if (n < 1 || n > TC_YPOINTS || m < 1 || m > GMM_MAX_TOPM) return cudaErrorInvalidValue;
-    if (m <= 4) return launch_assign_t<6>(s, X, n, D, K, mu, w2, c2, tb, rec, m, idx, resp, status);
-    return launch_assign_t<10>(s, X, n, D, K, mu, w2, c2, tb, rec, m, idx, resp, status);
+    if (m <= 4) return launch_assign_t<6>(s, X, n, D, K, mu, w2, c2, tb, rec, unc_rows, unc_count, m, idx, resp, status);
+    return launch_assign_t<10>(s, X, n, D, K, mu, w2, c2, tb, rec, unc_rows, unc_count, m, idx, resp, status);
 }
 
 }  // namespace fg

@@ -42,7 +42,7 @@ __device__ __forceinline__ float fast_ex2(float x) {
 template <typename ACC>
 __device__ __forceinline__ void tile_quadratic(TileSmem& sm, const float* __restrict__ X, int64_t row0, int64_t n,
                                                int D, const float* __restrict__ mu, const float* __restrict__ w2,
-                                               int k0, int K, ACC (&q)[4][4]) {
+                                               int k0, int K, ACC (&q)[4][4], const int32_t* __restrict__ gather = nullptr) {
     constexpr bool HP = sizeof(ACC) == 8;
     const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
 #pragma unroll
@@ -59,11 +59,12 @@ __device__ __forceinline__ void tile_quadratic(TileSmem& sm, const float* __rest
 #pragma unroll
         for (int j = 0; j < 2; ++j) {
             const int e4 = tid + j * NTHREADS, r = e4 >> 3, d = d0 + (e4 & 7) * 4;
-            const int64_t row = row0 + r;
+            const int64_t slot = row0 + r;
+            const int64_t row = (gather && slot < n) ? (int64_t)__ldg(gather + slot) : slot;     // gather: the tile's rows are X[gather[slot]], slot < n
             const int k = k0 + r;
             px[j] = pm[j] = pw[j] = make_float4(0.f, 0.f, 0.f, 0.f);
             if (vec && d + 4 <= D) {
-                if (row < n) px[j] = __ldg(reinterpret_cast<const float4*>(X + row * D + d));
+                if (slot < n) px[j] = __ldg(reinterpret_cast<const float4*>(X + row * D + d));
                 if (k < K) {
                     pm[j] = __ldg(reinterpret_cast<const float4*>(mu + (size_t)k * D + d));
                     pw[j] = __ldg(reinterpret_cast<const float4*>(w2 + (size_t)k * D + d));
@@ -73,7 +74,7 @@ __device__ __forceinline__ void tile_quadratic(TileSmem& sm, const float* __rest
 #pragma unroll
                 for (int t = 0; t < 4; ++t)
                     if (d + t < D) {
-                        if (row < n) xv[t] = __ldg(X + row * D + d + t);
+                        if (slot < n) xv[t] = __ldg(X + row * D + d + t);
                         if (k < K) {
                             mv[t] = __ldg(mu + (size_t)k * D + d + t);
                             wv[t] = __ldg(w2 + (size_t)k * D + d + t);
@@ -156,10 +157,16 @@ __global__ void __launch_bounds__(NTHREADS)
 lse_kernel(const float* __restrict__ X, int64_t n, int D, int K, const float* __restrict__ mu,
            const float* __restrict__ w2, const double* __restrict__ c2, double* __restrict__ logZ2,
            double* __restrict__ llpart, int m_out, int32_t* __restrict__ idx_out, float* __restrict__ resp_out,
-           const int* __restrict__ run_if) {
+           const int* __restrict__ run_if, const int32_t* __restrict__ gather, const int* __restrict__ gather_count) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     // run_if: the launch does nothing unless run_if[0] != 0 (the tensor-core assignment covers the other case)
     if (run_if && run_if[0] == 0) return;
+    // gather: the points are X[gather[0 .. *gather_count)] (top-m outputs go to those rows); CTAs beyond the count leave
+    if (gather) {
+        const int64_t cnt = *gather_count;
+        n = cnt < n ? cnt : n;
+        if ((int64_t)blockIdx.x * TP >= n) return;
+    }
     TileSmem& sm = *reinterpret_cast<TileSmem*>(smem_raw);
     __shared__ double ll_s[TP];
     const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
@@ -178,7 +185,7 @@ lse_kernel(const float* __restrict__ X, int64_t n, int D, int K, const float* __
 
     for (int k0 = 0; k0 < K; k0 += TC) {
         ACC q[4][4];
-        tile_quadratic<ACC>(sm, X, row0, n, D, mu, w2, k0, K, q);
+        tile_quadratic<ACC>(sm, X, row0, n, D, mu, w2, k0, K, q, gather);
         ACC cv[4];
 #pragma unroll
         for (int b = 0; b < 4; ++b) {
@@ -249,6 +256,7 @@ lse_kernel(const float* __restrict__ X, int64_t n, int D, int K, const float* __
             ACC* cv = cand_v + tid * 16 * M;
             int* ci = cand_i + tid * 16 * M;
             const double lzp = lz_s[tid];
+            const int64_t out_row = gather ? (int64_t)__ldg(gather + row0 + tid) : row0 + tid;
             for (int j = 0; j < m_out; ++j) {
                 int best = -1;
                 for (int s = 0; s < 16 * M; ++s) {
@@ -262,8 +270,8 @@ lse_kernel(const float* __restrict__ X, int64_t n, int D, int K, const float* __
                     r = fast_ex2((float)((double)cv[best] - lzp));
                     ci[best] = -1;
                 }
-                idx_out[(row0 + tid) * m_out + j] = id;
-                resp_out[(row0 + tid) * m_out + j] = r;
+                idx_out[out_row * m_out + j] = id;
+                resp_out[out_row * m_out + j] = r;
             }
         }
     }
@@ -586,37 +594,39 @@ cudaError_t launch_lse_fp32(cudaStream_t s, const float* X, int64_t n, int D, in
                             const float* w2, const double* c2d, double* logZ2, double* llpart) {
     const unsigned blocks = (unsigned)((n + TP - 1) / TP);
     if (fp32_high_precision(D))
-        lse_kernel<0, double><<<blocks, NTHREADS, sizeof(TileSmem), s>>>(X, n, D, K, mu, w2, c2d, logZ2, llpart, 0, nullptr, nullptr, nullptr);
+        lse_kernel<0, double><<<blocks, NTHREADS, sizeof(TileSmem), s>>>(X, n, D, K, mu, w2, c2d, logZ2, llpart, 0, nullptr, nullptr, nullptr, nullptr, nullptr);
     else
-        lse_kernel<0, float><<<blocks, NTHREADS, sizeof(TileSmem), s>>>(X, n, D, K, mu, w2, c2d, logZ2, llpart, 0, nullptr, nullptr, nullptr);
+        lse_kernel<0, float><<<blocks, NTHREADS, sizeof(TileSmem), s>>>(X, n, D, K, mu, w2, c2d, logZ2, llpart, 0, nullptr, nullptr, nullptr, nullptr, nullptr);
     return cudaGetLastError();
 }
 
 template <int M, typename ACC>
 static cudaError_t launch_topm_t(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu,
-                                 const float* w2, const double* c2d, int m, int32_t* idx, float* resp, const int* run_if) {
+                                 const float* w2, const double* c2d, int m, int32_t* idx, float* resp, const int* run_if,
+                                 const int32_t* gather, const int* gather_count) {
     size_t smem = sizeof(TileSmem);
     const size_t need = (size_t)TP * 16 * M * (sizeof(ACC) + 4);
     if (need > smem) smem = need;
     cudaError_t e = cudaFuncSetAttribute(lse_kernel<M, ACC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     const unsigned blocks = (unsigned)((n + TP - 1) / TP);
-    lse_kernel<M, ACC><<<blocks, NTHREADS, smem, s>>>(X, n, D, K, mu, w2, c2d, nullptr, nullptr, m, idx, resp, run_if);
+    lse_kernel<M, ACC><<<blocks, NTHREADS, smem, s>>>(X, n, D, K, mu, w2, c2d, nullptr, nullptr, m, idx, resp, run_if, gather, gather_count);
     return cudaGetLastError();
 }
 
 cudaError_t launch_topm_fp32(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu,
-                             const float* w2, const double* c2d, int m, int32_t* idx, float* resp, const int* run_if) {
+                             const float* w2, const double* c2d, int m, int32_t* idx, float* resp, const int* run_if,
+                             const int32_t* gather, const int* gather_count) {
     if (fp32_high_precision(D)) {
-        if (m <= 1) return launch_topm_t<1, double>(s, X, n, D, K, mu, w2, c2d, m, idx, resp, run_if);
-        if (m <= 2) return launch_topm_t<2, double>(s, X, n, D, K, mu, w2, c2d, m, idx, resp, run_if);
-        if (m <= 4) return launch_topm_t<4, double>(s, X, n, D, K, mu, w2, c2d, m, idx, resp, run_if);
-        return launch_topm_t<8, double>(s, X, n, D, K, mu, w2, c2d, m, idx, resp, run_if);
+        if (m <= 1) return launch_topm_t<1, double>(s, X, n, D, K, mu, w2, c2d, m, idx, resp, run_if, gather, gather_count);
+        if (m <= 2) return launch_topm_t<2, double>(s, X, n, D, K, mu, w2, c2d, m, idx, resp, run_if, gather, gather_count);
+        if (m <= 4) return launch_topm_t<4, double>(s, X, n, D, K, mu, w2, c2d, m, idx, resp, run_if, gather, gather_count);
+        return launch_topm_t<8, double>(s, X, n, D, K, mu, w2, c2d, m, idx, resp, run_if, gather, gather_count);
     }
-    if (m <= 1) return launch_topm_t<1, float>(s, X, n, D, K, mu, w2, c2d, m, idx, resp, run_if);
-    if (m <= 2) return launch_topm_t<2, float>(s, X, n, D, K, mu, w2, c2d, m, idx, resp, run_if);
-    if (m <= 4) return launch_topm_t<4, float>(s, X, n, D, K, mu, w2, c2d, m, idx, resp, run_if);
-    return launch_topm_t<8, float>(s, X, n, D, K, mu, w2, c2d, m, idx, resp, run_if);
+    if (m <= 1) return launch_topm_t<1, float>(s, X, n, D, K, mu, w2, c2d, m, idx, resp, run_if, gather, gather_count);
+    if (m <= 2) return launch_topm_t<2, float>(s, X, n, D, K, mu, w2, c2d, m, idx, resp, run_if, gather, gather_count);
+    if (m <= 4) return launch_topm_t<4, float>(s, X, n, D, K, mu, w2, c2d, m, idx, resp, run_if, gather, gather_count);
+    return launch_topm_t<8, float>(s, X, n, D, K, mu, w2, c2d, m, idx, resp, run_if, gather, gather_count);
 }
 
 cudaError_t launch_mstep_fp32(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu,

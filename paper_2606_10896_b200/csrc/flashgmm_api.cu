@@ -642,15 +642,23 @@ int gmm_assign_topm(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const
         ctx->launches += 2;
         KL(launch_ill_cache_tc(ctx->stream, D, mu, ctx->w2(), ctx->c2(), tb));
         const int64_t piece = ctx->tc_piece;
-        const size_t need = (size_t)(N < piece ? N : piece) * assign_tc_record_bytes(m);
+        const int64_t cap = N < piece ? N : piece;
+        const size_t rec_bytes = align256((size_t)cap * assign_tc_record_bytes(m));
+        const size_t need = rec_bytes + align256((size_t)cap * sizeof(int32_t)) + 256;       // records, uncertain rows, their count
         CHECK(grow_buffer(ctx, &ctx->at_scratch, &ctx->at_scratch_bytes, need, "the assignment records"));
+        unsigned char* base = static_cast<unsigned char*>(ctx->at_scratch);
+        int32_t* unc_rows = reinterpret_cast<int32_t*>(base + rec_bytes);
+        int* unc_count = reinterpret_cast<int*>(base + need - 256);
         for (int64_t off = 0; off < N; off += piece) {
             const int64_t cnt = (N - off < piece) ? (N - off) : piece;
             CHECK(prof_begin(ctx));
             KL(launch_transform_tc(ctx->stream, X + off * D, cnt, D, tb));
-            KL(launch_assign_tc(ctx->stream, X + off * D, cnt, D, K, mu, ctx->w2(), ctx->c2(), tb,
-                                static_cast<float*>(ctx->at_scratch), m, idx + off * m, resp + off * m, &ctx->result()->status));
+            KL(launch_assign_tc(ctx->stream, X + off * D, cnt, D, K, mu, ctx->w2(), ctx->c2(), tb, reinterpret_cast<float*>(base),
+                                unc_rows, unc_count, m, idx + off * m, resp + off * m, &ctx->result()->status));
             ctx->launches++;
+            // the rows the refinement was not certain about: all K components exactly, by the FP32 tile kernel
+            KL(launch_topm_fp32(ctx->stream, X + off * D, cnt, D, K, mu, ctx->w2(), ctx->c2d(), m, idx + off * m, resp + off * m,
+                                nullptr, unc_rows, unc_count));
             CHECK(prof_end(ctx));
         }
         run_fp32_if = tb.flags + 3;

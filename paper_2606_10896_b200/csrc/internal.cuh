@@ -36,10 +36,12 @@ cudaError_t launch_lse_fp32(cudaStream_t s, const float* X, int64_t n, int D, in
 cudaError_t launch_mstep_fp32(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu,
                               const float* w2, const double* c2d, const double* logZ2, float* partials,
                               const Fp32Plan& plan);
-// run_if: NULL, or a device flag: the kernel does nothing unless run_if[0] != 0
+// run_if: NULL, or a device flag: the kernel does nothing unless run_if[0] != 0.
+// gather: NULL, or device row indices: the points are X[gather[0 .. min(n, *gather_count))], and the outputs go to those
+// rows of idx / resp (n then bounds the number of gathered points, and sizes the grid).
 cudaError_t launch_topm_fp32(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu,
                              const float* w2, const double* c2d, int m, int32_t* idx, float* resp,
-                             const int* run_if = nullptr);
+                             const int* run_if = nullptr, const int32_t* gather = nullptr, const int* gather_count = nullptr);
 
 // ---- shared by all paths -------------------------------------------------------------------------------------
 // stats (+)= sum over `splits` partial blocks, fixed order, float64.  Partial layout: [splits][K + 2*K*D] floats,

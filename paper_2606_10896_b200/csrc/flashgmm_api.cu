@@ -94,6 +94,8 @@ struct gmm_ctx {
     void* km_scratch = nullptr;      // k-means step: list offsets, per-segment float64 sums
     void* at_scratch = nullptr;      // tensor-core assignment: candidate records of one piece of points
     size_t at_scratch_bytes = 0;
+    void* km_unit = nullptr;         // k-means step on the tensor path: var = 1 [K x D], pi = 1 / K [K]
+    size_t km_unit_bytes = 0;
     size_t km_scratch_bytes = 0;
     size_t pl_scratch_bytes = 0;
     bool capPlanes = false;    // the scratch layout in force includes the tensor path's planes of Y
@@ -412,6 +414,7 @@ int gmm_destroy(gmm_ctx* ctx) {
     if (ctx->pl_scratch) cudaFree(ctx->pl_scratch);
     if (ctx->km_scratch) cudaFree(ctx->km_scratch);
     if (ctx->at_scratch) cudaFree(ctx->at_scratch);
+    if (ctx->km_unit) cudaFree(ctx->km_unit);
     if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
     if (ctx->ev_created)
         for (int i = 0; i < EVENT_POOL; ++i) {
@@ -615,6 +618,11 @@ namespace {
 int grow_buffer(gmm_ctx* ctx, void** buf, size_t* have, size_t need, const char* what);
 }
 
+namespace {
+int assign_topm_impl(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const float* pi, const float* mu,
+                     const float* var, int m, int32_t* idx, float* resp);
+}
+
 int gmm_assign_topm(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const float* pi, const float* mu,
                     const float* var, int m, int32_t* idx, float* resp) {
     CHECK(check_shape(ctx, N, D, K));
@@ -627,6 +635,13 @@ int gmm_assign_topm(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const
     if (m < 1 || m > K || m > GMM_MAX_TOPM) return fail(ctx, GMM_EINVAL, "m must be in [1, min(K, %d)] (got %d)", GMM_MAX_TOPM, m);
     DeviceGuard g(ctx->device);
     CHECK(ensure_scratch(ctx, D, K));
+    return assign_topm_impl(ctx, X, N, D, K, pi, mu, var, m, idx, resp);
+}
+
+namespace {
+// The assignment pass proper (arguments checked, scratch in place); also the nearest-centroid search of the k-means step.
+int assign_topm_impl(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const float* pi, const float* mu,
+                     const float* var, int m, int32_t* idx, float* resp) {
     CU(cudaMemsetAsync(&ctx->result()->status, 0, sizeof(int), ctx->stream));
     KL(launch_prepare_fp32(ctx->stream, D, K, pi, mu, var, ctx->w2(), ctx->c2(), ctx->c2d(), &ctx->result()->status));
     // Tensor-core assignment where the E+M step would take the tensor path too.  Ill-conditioned components are evaluated
@@ -670,6 +685,7 @@ int gmm_assign_topm(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const
     ctx->last_path = tensor ? GMM_PATH_TENSOR : GMM_PATH_FP32;
     return GMM_OK;
 }
+}  // namespace
 
 int gmm_tensor_path_supports(int D, int K) { return tc_supports(D, K) ? 1 : 0; }
 
@@ -769,12 +785,23 @@ int gmm_kmeans_step(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const
     CHECK(grow_buffer(ctx, &ctx->pl_scratch, &ctx->pl_scratch_bytes, pl_scratch_bytes(K), "the posting-list counters"));
     CHECK(grow_buffer(ctx, &ctx->km_scratch, &ctx->km_scratch_bytes, km_scratch_bytes(D, K), "the k-means partial sums"));
     // nearest centroid = top-1 component of a unit-variance, equal-weight mixture
-    KL(launch_kmeans_unit_params(ctx->stream, D, K, ctx->w2(), ctx->c2d()));
     float* resp = reinterpret_cast<float*>(work);                 // [N], not used afterwards except as the builder's input
     int32_t* items = work + N;                                    // [N]
-    for (int64_t off = 0; off < N; off += SUPER_TILE) {
-        const int64_t cnt = (N - off < SUPER_TILE) ? (N - off) : SUPER_TILE;
-        KL(launch_topm_fp32(ctx->stream, X + off * D, cnt, D, K, centroids, ctx->w2(), ctx->c2d(), 1, assign + off, resp + off));
+    const bool tensor = ctx->capPlanes && ctx->lay.tc && ctx->path != GMM_PATH_FP32;
+    if (tensor) {
+        // through the assignment pass of the tensor path, with that mixture written out: pi = 1 / K, var = 1
+        const size_t KD = (size_t)K * D;
+        CHECK(grow_buffer(ctx, &ctx->km_unit, &ctx->km_unit_bytes, (KD + (size_t)K) * sizeof(float), "the unit mixture of the k-means step"));
+        float* var_u = static_cast<float*>(ctx->km_unit);
+        float* pi_u = var_u + KD;
+        KL(launch_kmeans_unit_mixture(ctx->stream, D, K, pi_u, var_u));
+        CHECK(assign_topm_impl(ctx, X, N, D, K, pi_u, centroids, var_u, 1, assign, resp));
+    } else {
+        KL(launch_kmeans_unit_params(ctx->stream, D, K, ctx->w2(), ctx->c2d()));
+        for (int64_t off = 0; off < N; off += SUPER_TILE) {
+            const int64_t cnt = (N - off < SUPER_TILE) ? (N - off) : SUPER_TILE;
+            KL(launch_topm_fp32(ctx->stream, X + off * D, cnt, D, K, centroids, ctx->w2(), ctx->c2d(), 1, assign + off, resp + off));
+        }
     }
     // the points of every cluster in ascending order, then fixed-order float64 sums
     KL(launch_posting_lists(ctx->stream, assign, resp, N, 1, K, 1.0f, 1, ctx->pl_scratch, km_offsets(ctx->km_scratch), items));
@@ -787,7 +814,7 @@ int gmm_kmeans_step(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const
     CU(cudaMemcpyAsync(&v, &ctx->result()->ll[slot], sizeof(double), cudaMemcpyDeviceToHost, ctx->stream));
     CU(cudaStreamSynchronize(ctx->stream));
     if (inertia) *inertia = v;
-    ctx->last_path = GMM_PATH_FP32;
+    ctx->last_path = tensor ? GMM_PATH_TENSOR : GMM_PATH_FP32;
     return GMM_OK;
 }
 

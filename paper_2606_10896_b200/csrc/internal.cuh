@@ -69,6 +69,8 @@ size_t km_scratch_bytes(int D, int K);
 int64_t* km_offsets(void* scratch);                     // [K + 1] inside the scratch: the posting-list offsets go here
 double* km_inertia_k(void* scratch, int D, int K);      // [K] per-cluster inertia, written by launch_kmeans_update
 cudaError_t launch_kmeans_unit_params(cudaStream_t s, int D, int K, float* w2, double* c2d);
+// pi [K] = 1 / K, var [K x D] = 1: the mixture whose top-1 component is the nearest centroid
+cudaError_t launch_kmeans_unit_mixture(cudaStream_t s, int D, int K, float* pi, float* var);
 cudaError_t launch_kmeans_update(cudaStream_t s, const float* X, int D, int K, const float* cent_in, const int32_t* items,
                                  void* scratch, float* cent_out, int64_t* counts);
 

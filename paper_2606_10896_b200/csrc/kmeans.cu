@@ -89,6 +89,20 @@ size_t km_scratch_bytes(int D, int K) {
     return ((size_t)K * S * D + (size_t)K * S + (size_t)K) * sizeof(double) + (size_t)(K + 1) * sizeof(int64_t);
 }
 
+namespace {
+__global__ void km_unit_mixture_kernel(size_t KD, int K, float* __restrict__ pi, float* __restrict__ var) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < KD) var[i] = 1.f;
+    if (i < (size_t)K) pi[i] = 1.f / (float)K;
+}
+}  // namespace
+
+cudaError_t launch_kmeans_unit_mixture(cudaStream_t s, int D, int K, float* pi, float* var) {
+    const size_t KD = (size_t)K * D;
+    km_unit_mixture_kernel<<<(unsigned)((KD + 255) / 256), 256, 0, s>>>(KD, K, pi, var);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_kmeans_unit_params(cudaStream_t s, int D, int K, float* w2, double* c2d) {
     const size_t KD = (size_t)K * D;
     km_unit_params_kernel<<<(unsigned)((KD + 255) / 256), 256, 0, s>>>(KD, K, w2, c2d);

@@ -1113,22 +1113,29 @@ __global__ void __launch_bounds__(128) tc_prepare_kernel(int D, int K, const flo
 }
 
 // Ascending list of the ill-conditioned components (illb > 0): flags[2] = their number, flags[3] = 1 when there are more
-// than TC_MAX_ILL of them (the assignment then runs on the FP32 kernels).  One block of 1024 threads, Kpad <= 1024.
+// than TC_MAX_ILL of them (the assignment then runs on the FP32 kernels).  One block of 1024 threads takes the components
+// 1024 at a time.
 __global__ void __launch_bounds__(1024) tc_ill_list_kernel(int Kpad, const float* __restrict__ illb, int* __restrict__ ill_list,
                                                            int* __restrict__ flags) {
     __shared__ int wcount[32];
-    const int k = threadIdx.x, lane = k & 31, w = k >> 5;
-    const bool is = k < Kpad && illb[k] > 0.f;
-    const unsigned b = __ballot_sync(0xffffffffu, is);
-    if (lane == 0) wcount[w] = __popc(b);
-    __syncthreads();
-    int before = 0, total = 0;
-    for (int j = 0; j < 32; ++j) {
-        if (j < w) before += wcount[j];
-        total += wcount[j];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    int done = 0;                                    // listed so far (the same in every thread)
+    for (int base = 0; base < Kpad; base += 1024) {
+        const int k = base + threadIdx.x;
+        const bool is = k < Kpad && illb[k] > 0.f;
+        const unsigned b = __ballot_sync(0xffffffffu, is);
+        __syncthreads();                             // the previous round's counts have been read
+        if (lane == 0) wcount[w] = __popc(b);
+        __syncthreads();
+        int before = 0, total = 0;
+        for (int j = 0; j < 32; ++j) {
+            if (j < w) before += wcount[j];
+            total += wcount[j];
+        }
+        if (is) ill_list[done + before + __popc(b & ((1u << lane) - 1u))] = k;
+        done += total;
     }
-    if (is) ill_list[before + __popc(b & ((1u << lane) - 1u))] = k;
-    if (k == 0) { flags[2] = total; flags[3] = total > TC_MAX_ILL ? 1 : 0; }
+    if (threadIdx.x == 0) { flags[2] = done; flags[3] = done > TC_MAX_ILL ? 1 : 0; }
 }
 
 // One thread per listed ill-conditioned component: its 8 dimensions of largest weight, in descending order of the weight.
@@ -1227,6 +1234,8 @@ void tc_set_test_hooks(int silent_rank, unsigned long long wait_limit_ns) {
 void tc_set_order(int o) { g_tc_order = o; }
 
 bool tc_supports(int D, int K) { return D >= 1 && D <= 128 && K >= 1 && K <= 1024; }
+// The assignment kernels walk over the components in chunks of 128 inside one CTA: no group of CTAs, so K may be larger.
+bool tc_assign_supports(int D, int K) { return D >= 1 && D <= 128 && K >= 1 && K <= TC_ASSIGN_MAX_K; }
 
 TcPlan tc_plan(int D, int K, int num_sms) {
     TcPlan pl;
@@ -1236,21 +1245,6 @@ TcPlan tc_plan(int D, int K, int num_sms) {
     if (pl.Q < 1) pl.Q = 1;
     pl.n_ks = (D + 7) / 8;
     return pl;
-}
-
-size_t tc_scratch_bytes(int D, int K) {
-    if (!tc_supports(D, K)) return 0;
-    const TcPlan pl = tc_plan(D, K, 160);
-    size_t b = 0;
-    b += (size_t)pl.CL * 128 * 128 * 4;                    // P_hi image
-    b += (size_t)pl.CL * 65536;                            // P_lo image
-    b += (size_t)pl.Kpad * 4 * 2 + 512;                    // t_k, c_k, s_d
-    b += (size_t)pl.Kpad * (512 * 2 + 8 + 4) + sizeof(TcIllCache);      // row-major P planes, (t_k, c_k) pairs, ill-conditioned components
-    b += (size_t)pl.Q * pl.Kpad * TC_PCOLS * 8;            // float64 partials
-    b += (size_t)pl.Q * 16;
-    b += 5 * (size_t)pl.Q * 4 * pl.CL * 64 * 16;           // exchange slots
-    b += 2 * TC_YPLANE_BYTES;                              // fp16 planes of Y for one launch
-    return b + 8 * 256;
 }
 
 cudaError_t launch_prepare_tc(cudaStream_t s, int D, int K, const float* pi, const float* mu, const float* var,

@@ -11,6 +11,7 @@ constexpr int TC_BN = 64;            // points per tile
 constexpr int TC_FLUSH = 64;         // tiles between flushes of the TMEM accumulators into float64 partials (even)
 constexpr float TC_RSCALE = 4096.f;  // responsibilities are scaled by this power of two before the fp16 split
 constexpr int TC_PCOLS = 258;        // columns of a partial row: 256 statistics columns + N_k of each softmax group
+constexpr int TC_ASSIGN_MAX_K = 4096;  // the tensor-core assignment takes up to this many components (the E+M tile kernel: 1024)
 constexpr int TC_MAX_ILL = 256;       // ill-conditioned components the tensor-core assignment evaluates exactly for every point
 constexpr int64_t TC_YPOINTS = 1 << 19;   // points per launch of the tile kernel: capacity of the fp16 planes of Y in scratch
 constexpr size_t TC_YPLANE_BYTES = (size_t)TC_YPOINTS * 512;   // one plane: 256 fp16 values per point
@@ -52,13 +53,13 @@ struct TcBuffers {
     TcIllCache* ill_cache;    // filled by launch_ill_cache_tc
 };
 
-bool tc_supports(int D, int K);
+bool tc_supports(int D, int K);          // the E+M tile kernel
+bool tc_assign_supports(int D, int K);   // the assignment kernels (a superset)
 void tc_set_order(int o);   // MMA issue order: 0 = pairs E E M M, 1 = interleaved M(i) E(i+2), 2 = whichever of E(i+2), M(i+1) is ready first (default)
 // Time-out test: CTA `silent_rank` of group 0 never publishes its exchange slot for tile 0 (-1: off), and every device-side
 // wait gives up after wait_limit_ns (0: the default 2 s).  Process-wide, like tc_set_order.
 void tc_set_test_hooks(int silent_rank, unsigned long long wait_limit_ns);
 TcPlan tc_plan(int D, int K, int num_sms);
-size_t tc_scratch_bytes(int D, int K);
 cudaError_t tc_max_clusters(int D, int K, int* out);
 cudaError_t launch_prepare_tc(cudaStream_t s, int D, int K, const float* pi, const float* mu, const float* var,
                               const TcBuffers& tb, float cond_limit, int* status, bool ill_list = false);

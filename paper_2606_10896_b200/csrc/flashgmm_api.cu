@@ -46,7 +46,7 @@ ScratchLayout scratch_layout(int D, int K, bool planes) {
     L.llpart = take((size_t)(SUPER_TILE / FP32_TILE_P) * 8);
     L.result = take(sizeof(DevResult));
     L.stats = take(((size_t)K + 2 * KD) * 8);
-    L.tc = tc_supports(D, K);
+    L.tc = tc_assign_supports(D, K);           // the assignment kernels' shapes include the E+M tile kernel's
     L.tc_phi = L.tc_plo = L.tc_tk = L.tc_ck = L.tc_sd = L.tc_kap = L.tc_illb = L.tc_flags = L.tc_xg = L.tc_xl = L.tc_partial = L.tc_llpart = L.tc_yhi = L.tc_ylo = L.tc_phirm = L.tc_plorm = L.tc_tkck = L.tc_illlist = L.tc_illcache = 0;
     L.tc_partial_bytes = 0;
     if (L.tc) {
@@ -59,11 +59,13 @@ ScratchLayout scratch_layout(int D, int K, bool planes) {
         L.tc_kap = take(128 * 4);
         L.tc_illb = take((size_t)pl.Kpad * 4);
         L.tc_flags = take(16);
-        L.tc_xg = take((size_t)pl.Q * 4 * pl.CL * 64 * 16);
-        L.tc_xl = take((size_t)pl.Q * 4 * pl.CL * 256 * 16);
-        L.tc_partial_bytes = (size_t)pl.Q * pl.Kpad * TC_PCOLS * 8;
-        L.tc_partial = take(L.tc_partial_bytes);
-        L.tc_llpart = take((size_t)pl.Q * 16);
+        if (tc_supports(D, K)) {                // what only the E+M tile kernel needs
+            L.tc_xg = take((size_t)pl.Q * 4 * pl.CL * 64 * 16);
+            L.tc_xl = take((size_t)pl.Q * 4 * pl.CL * 256 * 16);
+            L.tc_partial_bytes = (size_t)pl.Q * pl.Kpad * TC_PCOLS * 8;
+            L.tc_partial = take(L.tc_partial_bytes);
+            L.tc_llpart = take((size_t)pl.Q * 16);
+        }
         L.tc_phirm = take((size_t)pl.Kpad * 512);
         L.tc_plorm = take((size_t)pl.Kpad * 512);
         L.tc_tkck = take((size_t)pl.Kpad * 8);
@@ -183,9 +185,11 @@ int fail(gmm_ctx* ctx, int code, const char* fmt, ...) {
 
 // The tensor path runs when it is forced or when AUTO picks it for the shape: only then are the planes of Y needed.
 bool auto_is_tensor(int D, int K) { return tc_supports(D, K) && K >= 64 && D >= 8; }
+// AUTO also uses the tensor-core assignment for the larger K that only the assignment kernels take: planes are needed then
+bool auto_wants_planes(int D, int K) { return tc_assign_supports(D, K) && K >= 64 && D >= 8; }
 
 int ensure_scratch(gmm_ctx* ctx, int D, int K) {
-    const bool planes = tc_supports(D, K) && (ctx->path == GMM_PATH_TENSOR || (ctx->path == GMM_PATH_AUTO && auto_is_tensor(D, K)));
+    const bool planes = tc_assign_supports(D, K) && (ctx->path == GMM_PATH_TENSOR || (ctx->path == GMM_PATH_AUTO && auto_wants_planes(D, K)));
     if (ctx->scratch && D == ctx->capD && K == ctx->capK && planes == ctx->capPlanes) return GMM_OK;
     const ScratchLayout L = scratch_layout(D, K, planes);
     if (L.total > ctx->scratch_bytes) {
@@ -209,7 +213,7 @@ int ensure_scratch(gmm_ctx* ctx, int D, int K) {
     ctx->capK = K;
     ctx->capPlanes = planes;
     ctx->tc_Q = 0;
-    if (L.tc) {
+    if (L.tc && tc_supports(D, K)) {
         int q = 0;
         CU(tc_max_clusters(D, K, &q));
         const TcPlan pl = tc_plan(D, K, 160);
@@ -693,7 +697,7 @@ int gmm_auto_path(int D, int K) { return auto_is_tensor(D, K) ? GMM_PATH_TENSOR 
 
 size_t gmm_scratch_bytes(int D, int K) {
     if (D < 1 || K < 1) return 0;
-    return scratch_layout(D, K, auto_is_tensor(D, K)).total;      // what a context in GMM_PATH_AUTO allocates
+    return scratch_layout(D, K, auto_wants_planes(D, K)).total;      // what a context in GMM_PATH_AUTO allocates
 }
 
 int64_t gmm_launch_count(const gmm_ctx* ctx) { return ctx ? ctx->launches : 0; }

@@ -379,10 +379,12 @@ def _topm_tensor_vs_oracle(fg, ctx, X, pi, mu, var, m, what, expect_path=None):
 
 
 @pytest.mark.parametrize("N,D,K,m", [(1500, 128, 1024, 4), (777, 30, 100, 2), (2000, 100, 200, 8), (300, 9, 1000, 1),
-                                     (4097, 64, 640, 3), (129, 128, 64, 4), (1000, 128, 1024, 1)])
+                                     (4097, 64, 640, 3), (129, 128, 64, 4), (1000, 128, 1024, 1),
+                                     (1500, 128, 4096, 4), (1100, 96, 2048, 2)])
 def test_topm_tensor_path_against_oracle(fg, ctx, N, D, K, m):
     """Tensor-core selection + exact refinement (Sections 4.2-4.3): several tiles of 128 points with a ragged tail, odd
-    numbers of 128-component chunks, dimensions that do not fill the 64-column atoms."""
+    numbers of 128-component chunks, dimensions that do not fill the 64-column atoms, and K beyond what the E+M tile
+    kernel takes (the paper's IVF sizes go up to K = 4096)."""
     X, pi, mu, var = _random_mixture(np.random.default_rng(N + D + K), N, D, K)
     _topm_tensor_vs_oracle(fg, ctx, X, pi, mu, var, m, f"tensor top-m N={N} D={D} K={K} m={m}")
 

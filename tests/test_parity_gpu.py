@@ -490,6 +490,24 @@ def test_config3_full_size_conservation_and_subsample(fg, ctx):
         got = _gpu_step(ctx, Xsub_d, pi0, mu0, var0)
         assert abs(got[3] - ref[3]) <= 1e-5 * abs(ref[3])
         assert_stats_close(len(rows), s, got[:3], ref[:3], f"path {path} config 3 subsample")
+    _full_size_topm_check(fg, ctx, X, spec, pi0, mu0, var0, "config 3, all rows, sampled")
+
+
+def _full_size_topm_check(fg, ctx, X, spec, pi0, mu0, var0, what, n_rows=3000):
+    """Top-4 assignment over ALL rows of X, as bench.py --assign-m 4 launches it, under the parameters one EM iteration
+    gives; a seeded sample of rows is compared with the oracle's assignment of those rows one by one."""
+    ctx.gmm_set_path(fg.GMM_PATH_AUTO)
+    pi, mu, var = _t(pi0), _t(mu0), _t(var0)
+    Nk, S1, S2, _ = ctx.gmm_em_step(X, pi, mu, var)
+    ctx.gmm_finalize(spec.N, Nk, S1, S2, spec.var_floor, pi, mu, var)
+    idx, resp = ctx.gmm_assign_topm(X, pi, mu, var, 4)
+    torch.cuda.synchronize()
+    assert ctx.gmm_last_path() == fg.GMM_PATH_TENSOR
+    assert int(idx.min()) >= 0 and int(idx.max()) < spec.K
+    rows = synth.subsample_rows(spec.N, n_rows, spec.seed + 17)
+    rows_d = torch.as_tensor(rows, device=DEV)
+    idx_r, resp_r, next_r = orc.topm(X[rows_d].cpu().numpy(), pi.cpu().numpy(), mu.cpu().numpy(), var.cpu().numpy(), 4)
+    assert_topm_matches(idx[rows_d].cpu().numpy(), resp[rows_d].cpu().numpy(), idx_r, resp_r, next_r, what=what)
 
 
 def _column_sums(X):
@@ -535,6 +553,7 @@ def test_config4_full_size_conservation_additivity_and_subsample(fg, ctx):
     np.testing.assert_allclose(a[0] + b[0], Nk, rtol=1e-6, atol=1e-6 * N / spec.K)
     np.testing.assert_allclose(a[2] + b[2], S2, rtol=2e-5, atol=1e-5 * N / spec.K)
     assert abs((a[3] + b[3]) - L) <= 1e-9 * abs(L)
+    _full_size_topm_check(fg, ctx, X, spec, pi0, mu0, var0, "config 4, all rows, sampled")
     # oracle on a seeded subsample, GPU re-run on the same rows
     rows = synth.subsample_rows(N, 50_000, spec.seed)
     Xsub_d = X[torch.as_tensor(rows, device=DEV)].contiguous()

@@ -41,8 +41,9 @@ def parse():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--path", default="auto", choices=["auto", "fp32", "tensor"])
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--assign-m", type=int, default=0,
-                    help="also time gmm_assign_topm with this m on the same X (after the EM steps; reported as 'assign_topm')")
+    ap.add_argument("--assign-m", type=int, default=4,
+                    help="also time gmm_assign_topm with this m on the same X (after the timed EM steps, outside their "
+                         "timed region; reported as 'assign_topm'); 0 skips it")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
 

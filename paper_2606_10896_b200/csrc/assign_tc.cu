@@ -14,14 +14,18 @@
 //                      buffer; two such buffers, one per softmax warpgroup, alternate.  A softmax thread keeps for its point
 //                      the running (max, sum) of the log-sum-exp and the LIST largest logits with their indices, and
 //                      writes one record per tile.
-//   assign_refine_kernel  one warp per point: merges the records of the two warpgroups, recomputes the LIST - 1 best
-//                      candidates EXACTLY (fp32 direct differences, the arithmetic of the FP32 path), corrects the
-//                      log-sum-exp by the difference between exact and approximate candidate terms, orders by the exact
-//                      values (ties to the smaller index) and writes the top m.  The selection is certain when the m-th
-//                      exact value clears the best non-candidate's approximate value by more than the error bound of the
-//                      approximation; otherwise (near ties, exact ties, fewer than m finite candidates, broad
+//   assign_refine_kernel  first one thread per point: it merges the records of the two warpgroups, and where a single
+//                      component matters (all others below 2^-21 of it) it writes the answer from the approximate values.
+//                      The other points are taken by a whole warp each: the candidates that matter (at most LIST - 1)
+//                      are recomputed EXACTLY (fp32 direct differences, the arithmetic of the FP32 path), the
+//                      log-sum-exp is corrected by the difference between exact and approximate candidate terms, the
+//                      exact values are ordered (ties to the smaller index) and the top m written.  That result is
+//                      certain when the m-th exact value clears the best value left outside by more than the error
+//                      bound of the approximation, and accurate when the terms that stayed approximate are a small part
+//                      of the log-sum-exp; otherwise (near ties, exact ties, fewer than m finite candidates, broad
 //                      posteriors) the row is put on a list, and the FP32 tile kernel evaluates the listed rows against
-//                      all K components afterwards.
+//                      all K components afterwards.  Ill-conditioned components take no part in the selection and are
+//                      evaluated exactly where a test on their 8 dimensions of largest weight does not rule them out.
 #include "internal.cuh"
 #include "em_tc.cuh"
 
@@ -395,7 +399,7 @@ struct PointRow {
 };
 
 #ifdef FLASHGMM_DEBUG
-__device__ unsigned long long g_refine_counts[4];     // sharp points, exact candidate evaluations, exact ill evaluations, full scans
+__device__ unsigned long long g_refine_counts[4];     // points answered by one thread, exact candidate evaluations, exact ill evaluations, rows left uncertain
 #define RCOUNT(i, v) do { if (lane == 0) atomicAdd(&g_refine_counts[i], (unsigned long long)(v)); } while (0)
 #else
 #define RCOUNT(i, v)
@@ -532,7 +536,6 @@ __device__ __forceinline__ void refine_point(const RefineArgs& g, const TcIllCac
     // others).
     float ev = NEG, ea = NEG, tmax = 0.f;
     int evaluated = 0;
-    const bool stopped = false;
     if (p >= 2 || (p == 1 && n_exact > 0)) {
         float qv[C];
         int kv[C];
@@ -572,7 +575,7 @@ __device__ __forceinline__ void refine_point(const RefineArgs& g, const TcIllCac
     // The first m come from the exact list, then from the unevaluated candidates in approximate order.
     bool certain = n_top + (nvalid - evaluated) >= m && (n_top >= m || nvalid <= C || next_a < matter || evaluated == 0);
     if (certain && n_top >= m)
-        certain = stopped || next_a == NEG || next_a < matter || top.value_at(m - 1) > next_a + ebound;
+        certain = next_a == NEG || next_a < matter || top.value_at(m - 1) > next_a + ebound;
     float M = fmaxf(m0, m1), S = 0.f;
     if (certain) {
         if (n_top > 0) M = fmaxf(M, top.v[0]);
@@ -616,7 +619,7 @@ __device__ __forceinline__ void refine_point(const RefineArgs& g, const TcIllCac
 
 // A warp takes 32 consecutive points.  First every lane looks at one point on its own: it merges the records of the two
 // warpgroups and, if only one component matters for the point (the second best approximate value lies 21 + the error
-// bound below the best, and no ill-conditioned component passes the 8-dimension test), writes the answer straight from
+// bound below the best, and no ill-conditioned component passes the test on its 8 decisive dimensions), writes the answer straight from
 // the approximate values: the best responsibility is 1 - (the rest), the others are below 6e-8.  The points that are
 // left are then taken one after the other by the whole warp (refine_point).
 template <int LIST, int MAXM>

@@ -7,7 +7,11 @@
 //   registers across ALL its tiles (Algorithm 1, Step 2) -- the accumulators leave the SM once, as a per-CTA
 //   partial; there are no atomics.
 // The arithmetic is in the log2 domain: w2 = (log2 e / 2) / var, c2 = log2 e * (log pi - 1/2 sum_d log(2 pi var)),
-// log2 z = c2 - sum_d w2 (x - mu)^2, so the exponential is a bare ex2.
+// log2 z = c2 - sum_d w2 (x - mu)^2, so the exponential is a bare ex2.  A term w2 (x - mu)^2 is formed as t^2 with
+// t = (x - g) sqrt(w2) - (mu - g) sqrt(w2): one FMA for t (the second product is prepared when the tile is staged) and
+// one for the sum, instead of a subtraction, a product and an FMA.  g is a per-dimension centre (the mean of the
+// component means): with it both products are of the size of the data's spread, not of its distance from the origin, so
+// the rounding of the prepared product stays as harmless as that of the direct difference.
 #include "internal.cuh"
 #include <math_constants.h>
 #include <stdint.h>
@@ -35,14 +39,15 @@ __device__ __forceinline__ float fast_ex2(float x) {
 }
 
 // q[a][b] = sum_d w2[k0 + 4 tx + b][d] * (X[row0 + 4 ty + a][d] - mu[k0 + 4 tx + b][d])^2
-// Rows >= n and components >= K are staged as zeros (w2 = 0 -> contributes nothing).
+// Rows >= n and components >= K are staged as zeros (w2 = 0 -> contributes nothing).  g: per-dimension centre (may be NULL = 0).
 // ACC = float: one fp32 accumulation chain over D (D <= 128: a few 1e-6 of error).  ACC = double: each 32-dimension
 // chunk is summed in fp32 and the chunk sums are added in float64, which keeps long chains (D = 768: |q| ~ 1000 in the
 // log2 domain) from drowning the responsibilities in rounding noise.
 template <typename ACC>
 __device__ __forceinline__ void tile_quadratic(TileSmem& sm, const float* __restrict__ X, int64_t row0, int64_t n,
                                                int D, const float* __restrict__ mu, const float* __restrict__ w2,
-                                               int k0, int K, ACC (&q)[4][4], const int32_t* __restrict__ gather = nullptr) {
+                                               int k0, int K, ACC (&q)[4][4], const float* __restrict__ g,
+                                               const int32_t* __restrict__ gather = nullptr) {
     constexpr bool HP = sizeof(ACC) == 8;
     const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
 #pragma unroll
@@ -53,8 +58,8 @@ __device__ __forceinline__ void tile_quadratic(TileSmem& sm, const float* __rest
     // 128 bytes of one row) while the current 32 are being computed from shared memory, so the load latency is hidden
     // behind the arithmetic instead of being exposed at every stage.
     const bool vec = (D % 4 == 0) && (((reinterpret_cast<uintptr_t>(X) | reinterpret_cast<uintptr_t>(mu) |
-                                        reinterpret_cast<uintptr_t>(w2)) & 15) == 0);
-    float4 px[2], pm[2], pw[2];
+                                        reinterpret_cast<uintptr_t>(w2) | reinterpret_cast<uintptr_t>(g)) & 15) == 0);
+    float4 px[2], pm[2], pw[2], pg[2];
     auto fetch = [&](int d0) {
 #pragma unroll
         for (int j = 0; j < 2; ++j) {
@@ -62,8 +67,9 @@ __device__ __forceinline__ void tile_quadratic(TileSmem& sm, const float* __rest
             const int64_t slot = row0 + r;
             const int64_t row = (gather && slot < n) ? (int64_t)__ldg(gather + slot) : slot;     // gather: the tile's rows are X[gather[slot]], slot < n
             const int k = k0 + r;
-            px[j] = pm[j] = pw[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+            px[j] = pm[j] = pw[j] = pg[j] = make_float4(0.f, 0.f, 0.f, 0.f);
             if (vec && d + 4 <= D) {
+                if (g) pg[j] = __ldg(reinterpret_cast<const float4*>(g + d));
                 if (slot < n) px[j] = __ldg(reinterpret_cast<const float4*>(X + row * D + d));
                 if (k < K) {
                     pm[j] = __ldg(reinterpret_cast<const float4*>(mu + (size_t)k * D + d));
@@ -71,9 +77,11 @@ __device__ __forceinline__ void tile_quadratic(TileSmem& sm, const float* __rest
                 }
             } else {
                 float xv[4] = {0.f, 0.f, 0.f, 0.f}, mv[4] = {0.f, 0.f, 0.f, 0.f}, wv[4] = {0.f, 0.f, 0.f, 0.f};
+                float gv[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
                 for (int t = 0; t < 4; ++t)
                     if (d + t < D) {
+                        if (g) gv[t] = __ldg(g + d + t);
                         if (slot < n) xv[t] = __ldg(X + row * D + d + t);
                         if (k < K) {
                             mv[t] = __ldg(mu + (size_t)k * D + d + t);
@@ -83,6 +91,7 @@ __device__ __forceinline__ void tile_quadratic(TileSmem& sm, const float* __rest
                 px[j] = make_float4(xv[0], xv[1], xv[2], xv[3]);
                 pm[j] = make_float4(mv[0], mv[1], mv[2], mv[3]);
                 pw[j] = make_float4(wv[0], wv[1], wv[2], wv[3]);
+                pg[j] = make_float4(gv[0], gv[1], gv[2], gv[3]);
             }
         }
     };
@@ -92,9 +101,13 @@ __device__ __forceinline__ void tile_quadratic(TileSmem& sm, const float* __rest
 #pragma unroll
         for (int j = 0; j < 2; ++j) {
             const int e4 = tid + j * NTHREADS, r = e4 >> 3, c = (e4 & 7) * 4;
-            sm.xs[c][r] = px[j].x; sm.xs[c + 1][r] = px[j].y; sm.xs[c + 2][r] = px[j].z; sm.xs[c + 3][r] = px[j].w;
-            sm.ms[c][r] = pm[j].x; sm.ms[c + 1][r] = pm[j].y; sm.ms[c + 2][r] = pm[j].z; sm.ms[c + 3][r] = pm[j].w;
-            sm.ws[c][r] = pw[j].x; sm.ws[c + 1][r] = pw[j].y; sm.ws[c + 2][r] = pw[j].z; sm.ws[c + 3][r] = pw[j].w;
+            // staged: x - g, -(mu - g) sqrt(w), sqrt(w)   (zero weight for padded components: t = 0)
+            const float sx = sqrtf(pw[j].x), sy = sqrtf(pw[j].y), sz = sqrtf(pw[j].z), sq = sqrtf(pw[j].w);
+            sm.xs[c][r] = px[j].x - pg[j].x; sm.xs[c + 1][r] = px[j].y - pg[j].y;
+            sm.xs[c + 2][r] = px[j].z - pg[j].z; sm.xs[c + 3][r] = px[j].w - pg[j].w;
+            sm.ms[c][r] = (pg[j].x - pm[j].x) * sx; sm.ms[c + 1][r] = (pg[j].y - pm[j].y) * sy;
+            sm.ms[c + 2][r] = (pg[j].z - pm[j].z) * sz; sm.ms[c + 3][r] = (pg[j].w - pm[j].w) * sq;
+            sm.ws[c][r] = sx; sm.ws[c + 1][r] = sy; sm.ws[c + 2][r] = sz; sm.ws[c + 3][r] = sq;
         }
         __syncthreads();
         if (d0 + DCH < D) fetch(d0 + DCH);
@@ -115,8 +128,8 @@ __device__ __forceinline__ void tile_quadratic(TileSmem& sm, const float* __rest
             for (int a = 0; a < 4; ++a)
 #pragma unroll
                 for (int b = 0; b < 4; ++b) {
-                    const float diff = xa[a] - mb[b];
-                    part[a][b] = fmaf(diff * diff, wb[b], part[a][b]);
+                    const float t = fmaf(xa[a], wb[b], mb[b]);
+                    part[a][b] = fmaf(t, t, part[a][b]);
                 }
         }
 #pragma unroll
@@ -155,9 +168,10 @@ struct TopList {
 template <int M, typename ACC>
 __global__ void __launch_bounds__(NTHREADS)
 lse_kernel(const float* __restrict__ X, int64_t n, int D, int K, const float* __restrict__ mu,
-           const float* __restrict__ w2, const double* __restrict__ c2, double* __restrict__ logZ2,
-           double* __restrict__ llpart, int m_out, int32_t* __restrict__ idx_out, float* __restrict__ resp_out,
-           const int* __restrict__ run_if, const int32_t* __restrict__ gather, const int* __restrict__ gather_count) {
+           const float* __restrict__ w2, const double* __restrict__ c2, const float* __restrict__ g,
+           double* __restrict__ logZ2, double* __restrict__ llpart, int m_out, int32_t* __restrict__ idx_out,
+           float* __restrict__ resp_out, const int* __restrict__ run_if, const int32_t* __restrict__ gather,
+           const int* __restrict__ gather_count) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     // run_if: the launch does nothing unless run_if[0] != 0 (the tensor-core assignment covers the other case)
     if (run_if && run_if[0] == 0) return;
@@ -185,7 +199,7 @@ lse_kernel(const float* __restrict__ X, int64_t n, int D, int K, const float* __
 
     for (int k0 = 0; k0 < K; k0 += TC) {
         ACC q[4][4];
-        tile_quadratic<ACC>(sm, X, row0, n, D, mu, w2, k0, K, q, gather);
+        tile_quadratic<ACC>(sm, X, row0, n, D, mu, w2, k0, K, q, g, gather);
         ACC cv[4];
 #pragma unroll
         for (int b = 0; b < 4; ++b) {
@@ -292,8 +306,8 @@ constexpr size_t MSTEP_SMEM = sizeof(TileSmem) + (size_t)TP * LDR * 4 + (size_t)
 template <typename ACC>
 __global__ void __launch_bounds__(NTHREADS, sizeof(ACC) == 4 ? 2 : 1)      // float logits: two CTAs per SM
 mstep_kernel(const float* __restrict__ X, int64_t n, int D, int K, const float* __restrict__ mu,
-             const float* __restrict__ w2, const double* __restrict__ c2, const double* __restrict__ logZ2,
-             float* __restrict__ partials) {
+             const float* __restrict__ w2, const double* __restrict__ c2, const float* __restrict__ g,
+             const double* __restrict__ logZ2, float* __restrict__ partials) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     TileSmem& sm = *reinterpret_cast<TileSmem*>(smem_raw);
     float* r_s = reinterpret_cast<float*>(smem_raw + sizeof(TileSmem));     // [TP][LDR]
@@ -321,7 +335,7 @@ mstep_kernel(const float* __restrict__ X, int64_t n, int D, int K, const float* 
     for (int64_t t = split; t < ntiles; t += nsplits) {
         const int64_t row0 = t * TP;
         ACC q[4][4];
-        tile_quadratic<ACC>(sm, X, row0, n, D, mu, w2, k0, K, q);
+        tile_quadratic<ACC>(sm, X, row0, n, D, mu, w2, k0, K, q, g);
 #pragma unroll
         for (int a = 0; a < 4; ++a) {
             const int64_t row = row0 + 4 * ty + a;
@@ -397,8 +411,8 @@ constexpr size_t MSTEP_WIDE_SMEM = sizeof(TileSmem) + (size_t)WT * TP * LDR * 4 
 
 __global__ void __launch_bounds__(NTHREADS, 2)
 mstep_wide_kernel(const float* __restrict__ X, int64_t n, int D, int K, const float* __restrict__ mu,
-                  const float* __restrict__ w2, const double* __restrict__ c2, const double* __restrict__ logZ2,
-                  double* __restrict__ partials) {
+                  const float* __restrict__ w2, const double* __restrict__ c2, const float* __restrict__ g,
+                  const double* __restrict__ logZ2, double* __restrict__ partials) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     TileSmem& sm = *reinterpret_cast<TileSmem*>(smem_raw);
     float* r_all = reinterpret_cast<float*>(smem_raw + sizeof(TileSmem));   // [WT][TP][LDR]
@@ -431,7 +445,7 @@ mstep_wide_kernel(const float* __restrict__ X, int64_t n, int D, int K, const fl
             ++nb;
             const int64_t row0 = t * TP;
             double q[4][4];
-            tile_quadratic<double>(sm, X, row0, n, D, mu, w2, k0, K, q);
+            tile_quadratic<double>(sm, X, row0, n, D, mu, w2, k0, K, q, g);
             float* r_s = r_all + w * TP * LDR;
 #pragma unroll
             for (int a = 0; a < 4; ++a) {
@@ -511,8 +525,17 @@ mstep_wide_kernel(const float* __restrict__ X, int64_t n, int D, int K, const fl
 // One block per component: w2 = (log2 e / 2) / var, c2 = log2 e (log pi - 1/2 sum_d log(2 pi var)), in float64.
 __global__ void prepare_fp32_kernel(int D, int K, const float* __restrict__ pi, const float* __restrict__ mu,
                                     const float* __restrict__ var, float* __restrict__ w2, float* __restrict__ c2,
-                                    double* __restrict__ c2d, int* __restrict__ status) {
+                                    double* __restrict__ c2d, int* __restrict__ status, float* __restrict__ g_small) {
     const int k = blockIdx.x;
+    // small problems (launch-bound): block 0 also forms the centre of the means, which saves a launch
+    if (g_small && k == 0) {
+        for (int d = threadIdx.x; d < D; d += blockDim.x) {
+            double s = 0.0;
+            for (int kk = 0; kk < K; ++kk) s += (double)mu[(size_t)kk * D + d];
+            const float c = (float)(s / (double)K);
+            g_small[d] = isfinite(c) ? c : 0.f;
+        }
+    }
     __shared__ double red[128];
     double s = 0.0;
     int bad = 0;
@@ -540,6 +563,26 @@ __global__ void prepare_fp32_kernel(int D, int K, const float* __restrict__ pi, 
         c2d[k] = cd;
     }
     if (bad) atomicOr(status, bad);
+}
+
+// g[d] = mean over the components of mu[k][d]: the centre the tile routine subtracts from points and means.  A block takes
+// 32 dimensions; its 8 warps sum every 8th component in float64 and the 8 partial sums are added in a fixed order.  A
+// non-finite mean (reported through the status word by prepare_fp32_kernel) gives centre 0.
+__global__ void __launch_bounds__(256) center_fp32_kernel(int D, int K, const float* __restrict__ mu, float* __restrict__ g) {
+    __shared__ double part[8][32];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int d = blockIdx.x * 32 + lane;
+    double s = 0.0;
+    if (d < D)
+        for (int k = w; k < K; k += 8) s += (double)mu[(size_t)k * D + d];
+    part[w][lane] = s;
+    __syncthreads();
+    if (w == 0 && d < D) {
+        double t = 0.0;
+        for (int j = 0; j < 8; ++j) t += part[j][lane];
+        const float c = (float)(t / (double)K);
+        g[d] = isfinite(c) ? c : 0.f;
+    }
 }
 
 }  // namespace
@@ -581,56 +624,64 @@ size_t fp32_partial_floats(int D, int K) {
     return (size_t)p.splits * ((size_t)K + 2 * (size_t)K * D) * (p.wide ? 2 : 1);
 }
 
-cudaError_t launch_prepare_fp32(cudaStream_t s, int D, int K, const float* pi, const float* mu, const float* var,
-                                float* w2, float* c2, double* c2d, int* status) {
-    prepare_fp32_kernel<<<K, 128, 0, s>>>(D, K, pi, mu, var, w2, c2, c2d, status);
+cudaError_t launch_center_fp32(cudaStream_t s, int D, int K, const float* mu, float* g) {
+    center_fp32_kernel<<<(unsigned)((D + 31) / 32), 256, 0, s>>>(D, K, mu, g);
     return cudaGetLastError();
+}
+
+cudaError_t launch_prepare_fp32(cudaStream_t s, int D, int K, const float* pi, const float* mu, const float* var,
+                                float* w2, float* c2, double* c2d, float* g, int* status) {
+    const bool small = g && (size_t)K * D <= ((size_t)1 << 12);
+    prepare_fp32_kernel<<<K, 128, 0, s>>>(D, K, pi, mu, var, w2, c2, c2d, status, small ? g : nullptr);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess || !g || small) return e;
+    return launch_center_fp32(s, D, K, mu, g);
 }
 
 // Logits are carried in float64 when the accumulation over D is long.
 static inline bool fp32_high_precision(int D) { return D > 128; }
 
 cudaError_t launch_lse_fp32(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu,
-                            const float* w2, const double* c2d, double* logZ2, double* llpart) {
+                            const float* w2, const double* c2d, const float* g, double* logZ2, double* llpart) {
     const unsigned blocks = (unsigned)((n + TP - 1) / TP);
     if (fp32_high_precision(D))
-        lse_kernel<0, double><<<blocks, NTHREADS, sizeof(TileSmem), s>>>(X, n, D, K, mu, w2, c2d, logZ2, llpart, 0, nullptr, nullptr, nullptr, nullptr, nullptr);
+        lse_kernel<0, double><<<blocks, NTHREADS, sizeof(TileSmem), s>>>(X, n, D, K, mu, w2, c2d, g, logZ2, llpart, 0, nullptr, nullptr, nullptr, nullptr, nullptr);
     else
-        lse_kernel<0, float><<<blocks, NTHREADS, sizeof(TileSmem), s>>>(X, n, D, K, mu, w2, c2d, logZ2, llpart, 0, nullptr, nullptr, nullptr, nullptr, nullptr);
+        lse_kernel<0, float><<<blocks, NTHREADS, sizeof(TileSmem), s>>>(X, n, D, K, mu, w2, c2d, g, logZ2, llpart, 0, nullptr, nullptr, nullptr, nullptr, nullptr);
     return cudaGetLastError();
 }
 
 template <int M, typename ACC>
 static cudaError_t launch_topm_t(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu,
-                                 const float* w2, const double* c2d, int m, int32_t* idx, float* resp, const int* run_if,
-                                 const int32_t* gather, const int* gather_count) {
+                                 const float* w2, const double* c2d, const float* g, int m, int32_t* idx, float* resp,
+                                 const int* run_if, const int32_t* gather, const int* gather_count) {
     size_t smem = sizeof(TileSmem);
     const size_t need = (size_t)TP * 16 * M * (sizeof(ACC) + 4);
     if (need > smem) smem = need;
     cudaError_t e = cudaFuncSetAttribute(lse_kernel<M, ACC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     const unsigned blocks = (unsigned)((n + TP - 1) / TP);
-    lse_kernel<M, ACC><<<blocks, NTHREADS, smem, s>>>(X, n, D, K, mu, w2, c2d, nullptr, nullptr, m, idx, resp, run_if, gather, gather_count);
+    lse_kernel<M, ACC><<<blocks, NTHREADS, smem, s>>>(X, n, D, K, mu, w2, c2d, g, nullptr, nullptr, m, idx, resp, run_if, gather, gather_count);
     return cudaGetLastError();
 }
 
 cudaError_t launch_topm_fp32(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu,
-                             const float* w2, const double* c2d, int m, int32_t* idx, float* resp, const int* run_if,
-                             const int32_t* gather, const int* gather_count) {
+                             const float* w2, const double* c2d, const float* g, int m, int32_t* idx, float* resp,
+                             const int* run_if, const int32_t* gather, const int* gather_count) {
     if (fp32_high_precision(D)) {
-        if (m <= 1) return launch_topm_t<1, double>(s, X, n, D, K, mu, w2, c2d, m, idx, resp, run_if, gather, gather_count);
-        if (m <= 2) return launch_topm_t<2, double>(s, X, n, D, K, mu, w2, c2d, m, idx, resp, run_if, gather, gather_count);
-        if (m <= 4) return launch_topm_t<4, double>(s, X, n, D, K, mu, w2, c2d, m, idx, resp, run_if, gather, gather_count);
-        return launch_topm_t<8, double>(s, X, n, D, K, mu, w2, c2d, m, idx, resp, run_if, gather, gather_count);
+        if (m <= 1) return launch_topm_t<1, double>(s, X, n, D, K, mu, w2, c2d, g, m, idx, resp, run_if, gather, gather_count);
+        if (m <= 2) return launch_topm_t<2, double>(s, X, n, D, K, mu, w2, c2d, g, m, idx, resp, run_if, gather, gather_count);
+        if (m <= 4) return launch_topm_t<4, double>(s, X, n, D, K, mu, w2, c2d, g, m, idx, resp, run_if, gather, gather_count);
+        return launch_topm_t<8, double>(s, X, n, D, K, mu, w2, c2d, g, m, idx, resp, run_if, gather, gather_count);
     }
-    if (m <= 1) return launch_topm_t<1, float>(s, X, n, D, K, mu, w2, c2d, m, idx, resp, run_if, gather, gather_count);
-    if (m <= 2) return launch_topm_t<2, float>(s, X, n, D, K, mu, w2, c2d, m, idx, resp, run_if, gather, gather_count);
-    if (m <= 4) return launch_topm_t<4, float>(s, X, n, D, K, mu, w2, c2d, m, idx, resp, run_if, gather, gather_count);
-    return launch_topm_t<8, float>(s, X, n, D, K, mu, w2, c2d, m, idx, resp, run_if, gather, gather_count);
+    if (m <= 1) return launch_topm_t<1, float>(s, X, n, D, K, mu, w2, c2d, g, m, idx, resp, run_if, gather, gather_count);
+    if (m <= 2) return launch_topm_t<2, float>(s, X, n, D, K, mu, w2, c2d, g, m, idx, resp, run_if, gather, gather_count);
+    if (m <= 4) return launch_topm_t<4, float>(s, X, n, D, K, mu, w2, c2d, g, m, idx, resp, run_if, gather, gather_count);
+    return launch_topm_t<8, float>(s, X, n, D, K, mu, w2, c2d, g, m, idx, resp, run_if, gather, gather_count);
 }
 
 cudaError_t launch_mstep_fp32(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu,
-                              const float* w2, const double* c2d, const double* logZ2, float* partials,
+                              const float* w2, const double* c2d, const float* g, const double* logZ2, float* partials,
                               const Fp32Plan& plan) {
     if (plan.wide) {
         cudaError_t e = cudaFuncSetAttribute(mstep_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)MSTEP_WIDE_SMEM);
@@ -639,18 +690,18 @@ cudaError_t launch_mstep_fp32(cudaStream_t s, const float* X, int64_t n, int D, 
         e = cudaMemsetAsync(partials, 0, bytes, s);          // the kernel accumulates into its partials
         if (e != cudaSuccess) return e;
         dim3 wgrid(plan.comp_blocks, plan.splits, 1);
-        mstep_wide_kernel<<<wgrid, NTHREADS, MSTEP_WIDE_SMEM, s>>>(X, n, D, K, mu, w2, c2d, logZ2, reinterpret_cast<double*>(partials));
+        mstep_wide_kernel<<<wgrid, NTHREADS, MSTEP_WIDE_SMEM, s>>>(X, n, D, K, mu, w2, c2d, g, logZ2, reinterpret_cast<double*>(partials));
         return cudaGetLastError();
     }
     dim3 grid(plan.comp_blocks, plan.splits, plan.d_chunks);
     if (fp32_high_precision(D)) {
         cudaError_t e = cudaFuncSetAttribute(mstep_kernel<double>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)MSTEP_SMEM);
         if (e != cudaSuccess) return e;
-        mstep_kernel<double><<<grid, NTHREADS, MSTEP_SMEM, s>>>(X, n, D, K, mu, w2, c2d, logZ2, partials);
+        mstep_kernel<double><<<grid, NTHREADS, MSTEP_SMEM, s>>>(X, n, D, K, mu, w2, c2d, g, logZ2, partials);
     } else {
         cudaError_t e = cudaFuncSetAttribute(mstep_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)MSTEP_SMEM);
         if (e != cudaSuccess) return e;
-        mstep_kernel<float><<<grid, NTHREADS, MSTEP_SMEM, s>>>(X, n, D, K, mu, w2, c2d, logZ2, partials);
+        mstep_kernel<float><<<grid, NTHREADS, MSTEP_SMEM, s>>>(X, n, D, K, mu, w2, c2d, g, logZ2, partials);
     }
     return cudaGetLastError();
 }

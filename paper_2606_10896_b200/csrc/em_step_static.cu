@@ -31,7 +31,7 @@ struct StaticResult {
 };
 
 struct StaticLayout {
-    size_t w2, c2, c2d, logZ2, llpart, result, partials, total;
+    size_t w2, c2, c2d, center, logZ2, llpart, result, partials, total;
     int splits;
 };
 
@@ -48,6 +48,7 @@ StaticLayout static_layout(int D, int K) {
     L.w2 = take(KD * 4);
     L.c2 = take((size_t)K * 4);
     L.c2d = take((size_t)K * 8);
+    L.center = take((size_t)D * 4);
     L.logZ2 = take((size_t)STATIC_TILE * 8);
     L.llpart = take((size_t)(STATIC_TILE / FP32_TILE_P) * 8);
     L.result = take(sizeof(StaticResult));
@@ -104,6 +105,7 @@ extern "C" int gmm_em_step_static(int device, void* cuda_stream, const float* X,
     float* w2 = reinterpret_cast<float*>(base + L.w2);
     float* c2 = reinterpret_cast<float*>(base + L.c2);
     double* c2d = reinterpret_cast<double*>(base + L.c2d);
+    float* center = reinterpret_cast<float*>(base + L.center);
     double* logZ2 = reinterpret_cast<double*>(base + L.logZ2);
     double* llpart = reinterpret_cast<double*>(base + L.llpart);
     StaticResult* res = reinterpret_cast<StaticResult*>(base + L.result);
@@ -118,12 +120,12 @@ extern "C" int gmm_em_step_static(int device, void* cuda_stream, const float* X,
     SCU(cudaMemsetAsync(Nk, 0, (size_t)K * 8, s));
     SCU(cudaMemsetAsync(S1, 0, KD * 8, s));
     SCU(cudaMemsetAsync(S2, 0, KD * 8, s));
-    SCU(launch_prepare_fp32(s, D, K, pi, mu, var, w2, c2, c2d, &res->status));
+    SCU(launch_prepare_fp32(s, D, K, pi, mu, var, w2, c2, c2d, center, &res->status));
     for (int64_t off = 0; off < N; off += STATIC_TILE) {
         const int64_t cnt = (N - off < STATIC_TILE) ? (N - off) : STATIC_TILE;
         const float* Xs = X + off * D;
-        SCU(launch_lse_fp32(s, Xs, cnt, D, K, mu, w2, c2d, logZ2, llpart));
-        SCU(launch_mstep_fp32(s, Xs, cnt, D, K, mu, w2, c2d, logZ2, partials, plan));
+        SCU(launch_lse_fp32(s, Xs, cnt, D, K, mu, w2, c2d, center, logZ2, llpart));
+        SCU(launch_mstep_fp32(s, Xs, cnt, D, K, mu, w2, c2d, center, logZ2, partials, plan));
         SCU(launch_reduce_ll(s, llpart, (cnt + FP32_TILE_P - 1) / FP32_TILE_P, &res->ll, true));
         SCU(launch_reduce_partials(s, D, K, plan.splits, partials, Nk, S1, S2, true));
     }

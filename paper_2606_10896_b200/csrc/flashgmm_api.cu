@@ -27,7 +27,7 @@ constexpr int EVENT_POOL = 128;
 inline size_t align256(size_t b) { return (b + 255) & ~(size_t)255; }
 
 struct ScratchLayout {
-    size_t w2, c2, c2d, partials, logZ2, llpart, result, stats, total;
+    size_t w2, c2, c2d, center, partials, logZ2, llpart, result, stats, total;
     size_t tc_phi, tc_plo, tc_tk, tc_ck, tc_sd, tc_kap, tc_illb, tc_flags, tc_xg, tc_xl, tc_partial, tc_llpart, tc_partial_bytes, tc_yhi, tc_ylo, tc_phirm, tc_plorm, tc_tkck, tc_illlist, tc_illcache;
     bool tc;
 };
@@ -41,6 +41,7 @@ ScratchLayout scratch_layout(int D, int K, bool planes) {
     L.w2 = take(KD * 4);
     L.c2 = take((size_t)K * 4);
     L.c2d = take((size_t)K * 8);
+    L.center = take((size_t)D * 4);
     L.partials = take(fp32_partial_floats(D, K) * 4);
     L.logZ2 = take((size_t)SUPER_TILE * 8);
     L.llpart = take((size_t)(SUPER_TILE / FP32_TILE_P) * 8);
@@ -126,6 +127,7 @@ struct gmm_ctx {
     float* w2() const { return reinterpret_cast<float*>(scratch + lay.w2); }
     float* c2() const { return reinterpret_cast<float*>(scratch + lay.c2); }
     double* c2d() const { return reinterpret_cast<double*>(scratch + lay.c2d); }
+    float* center() const { return reinterpret_cast<float*>(scratch + lay.center); }     // per-dimension centre of the means
     float* partials() const { return reinterpret_cast<float*>(scratch + lay.partials); }
     double* logZ2() const { return reinterpret_cast<double*>(scratch + lay.logZ2); }
     double* llpart() const { return reinterpret_cast<double*>(scratch + lay.llpart); }
@@ -277,7 +279,8 @@ int prof_end(gmm_ctx* ctx) {
 int prepare_and_choose(gmm_ctx* ctx, int64_t N, int D, int K, const float* pi, const float* mu, const float* var,
                        int* path) {
     CU(cudaMemsetAsync(&ctx->result()->status, 0, sizeof(int), ctx->stream));
-    KL(launch_prepare_fp32(ctx->stream, D, K, pi, mu, var, ctx->w2(), ctx->c2(), ctx->c2d(), &ctx->result()->status));
+    KL(launch_prepare_fp32(ctx->stream, D, K, pi, mu, var, ctx->w2(), ctx->c2(), ctx->c2d(), ctx->center(), &ctx->result()->status));
+    if ((size_t)K * D > ((size_t)1 << 12)) ctx->launches++;      // but for tiny problems, the centre of the means is a launch of its own
     const bool tc_ok = ctx->lay.tc && ctx->tc_Q >= 1;
     const bool tc_auto = tc_ok && gmm_auto_path(D, K) == GMM_PATH_TENSOR;
     if (ctx->path == GMM_PATH_TENSOR && !tc_ok)
@@ -325,8 +328,8 @@ int accumulate_points(gmm_ctx* ctx, int path, const float* X, int64_t n, int D, 
         const int64_t cnt = (n - off < SUPER_TILE) ? (n - off) : SUPER_TILE;
         const float* Xs = X + off * D;
         CHECK(prof_begin(ctx));
-        KL(launch_lse_fp32(ctx->stream, Xs, cnt, D, K, mu, ctx->w2(), ctx->c2d(), ctx->logZ2(), ctx->llpart()));
-        KL(launch_mstep_fp32(ctx->stream, Xs, cnt, D, K, mu, ctx->w2(), ctx->c2d(), ctx->logZ2(), ctx->partials(), plan));
+        KL(launch_lse_fp32(ctx->stream, Xs, cnt, D, K, mu, ctx->w2(), ctx->c2d(), ctx->center(), ctx->logZ2(), ctx->llpart()));
+        KL(launch_mstep_fp32(ctx->stream, Xs, cnt, D, K, mu, ctx->w2(), ctx->c2d(), ctx->center(), ctx->logZ2(), ctx->partials(), plan));
         CHECK(prof_end(ctx));
         KL(launch_reduce_ll(ctx->stream, ctx->llpart(), (cnt + FP32_TILE_P - 1) / FP32_TILE_P, &ctx->result()->ll[slot], true));
         KL(launch_reduce_partials(ctx->stream, D, K, plan.splits, ctx->partials(), Nk, S1, S2, true));
@@ -647,7 +650,8 @@ namespace {
 int assign_topm_impl(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const float* pi, const float* mu,
                      const float* var, int m, int32_t* idx, float* resp) {
     CU(cudaMemsetAsync(&ctx->result()->status, 0, sizeof(int), ctx->stream));
-    KL(launch_prepare_fp32(ctx->stream, D, K, pi, mu, var, ctx->w2(), ctx->c2(), ctx->c2d(), &ctx->result()->status));
+    KL(launch_prepare_fp32(ctx->stream, D, K, pi, mu, var, ctx->w2(), ctx->c2(), ctx->c2d(), ctx->center(), &ctx->result()->status));
+    if ((size_t)K * D > ((size_t)1 << 12)) ctx->launches++;      // but for tiny problems, the centre of the means is a launch of its own
     // Tensor-core assignment where the E+M step would take the tensor path too.  Ill-conditioned components are evaluated
     // exactly for every point; parameters with more than TC_MAX_ILL of them (a flag written on the device by the
     // preparation kernels) go through the FP32 kernels instead: both sets of kernels are enqueued and each checks the
@@ -676,7 +680,7 @@ int assign_topm_impl(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, cons
                                 unc_rows, unc_count, m, idx + off * m, resp + off * m, &ctx->result()->status));
             ctx->launches++;
             // the rows the refinement was not certain about: all K components exactly, by the FP32 tile kernel
-            KL(launch_topm_fp32(ctx->stream, X + off * D, cnt, D, K, mu, ctx->w2(), ctx->c2d(), m, idx + off * m, resp + off * m,
+            KL(launch_topm_fp32(ctx->stream, X + off * D, cnt, D, K, mu, ctx->w2(), ctx->c2d(), ctx->center(), m, idx + off * m, resp + off * m,
                                 nullptr, unc_rows, unc_count));
             CHECK(prof_end(ctx));
         }
@@ -684,7 +688,7 @@ int assign_topm_impl(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, cons
     }
     for (int64_t off = 0; off < N; off += SUPER_TILE) {
         const int64_t cnt = (N - off < SUPER_TILE) ? (N - off) : SUPER_TILE;
-        KL(launch_topm_fp32(ctx->stream, X + off * D, cnt, D, K, mu, ctx->w2(), ctx->c2d(), m, idx + off * m, resp + off * m, run_fp32_if));
+        KL(launch_topm_fp32(ctx->stream, X + off * D, cnt, D, K, mu, ctx->w2(), ctx->c2d(), ctx->center(), m, idx + off * m, resp + off * m, run_fp32_if));
     }
     ctx->last_path = tensor ? GMM_PATH_TENSOR : GMM_PATH_FP32;
     return GMM_OK;
@@ -802,9 +806,10 @@ int gmm_kmeans_step(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const
         CHECK(assign_topm_impl(ctx, X, N, D, K, pi_u, centroids, var_u, 1, assign, resp));
     } else {
         KL(launch_kmeans_unit_params(ctx->stream, D, K, ctx->w2(), ctx->c2d()));
+        KL(launch_center_fp32(ctx->stream, D, K, centroids, ctx->center()));
         for (int64_t off = 0; off < N; off += SUPER_TILE) {
             const int64_t cnt = (N - off < SUPER_TILE) ? (N - off) : SUPER_TILE;
-            KL(launch_topm_fp32(ctx->stream, X + off * D, cnt, D, K, centroids, ctx->w2(), ctx->c2d(), 1, assign + off, resp + off));
+            KL(launch_topm_fp32(ctx->stream, X + off * D, cnt, D, K, centroids, ctx->w2(), ctx->c2d(), ctx->center(), 1, assign + off, resp + off));
         }
     }
     // the points of every cluster in ascending order, then fixed-order float64 sums

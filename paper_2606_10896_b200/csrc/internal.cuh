@@ -27,20 +27,24 @@ Fp32Plan fp32_plan(int D, int K);
 size_t fp32_partial_floats(int D, int K);   // floats in the per-CTA partial buffer
 
 // ---- FP32 (CUDA-core) path -----------------------------------------------------------------------------------
+// g [D] (may be NULL): receives the per-dimension centre of the means (launch_center_fp32), which the kernels below take
 cudaError_t launch_prepare_fp32(cudaStream_t s, int D, int K, const float* pi, const float* mu, const float* var,
-                                float* w2, float* c2, double* c2d, int* status);
+                                float* w2, float* c2, double* c2d, float* g, int* status);
+cudaError_t launch_center_fp32(cudaStream_t s, int D, int K, const float* mu, float* g);
 // log2-domain log Z of n points -> logZ2[n]; per-block float64 partial log-likelihoods -> llpart[ceil(n/64)]
 // c2d: the per-component constants in float64; logZ2: float64 (the kernels carry logits in float64 when D > 128)
+// g: the per-dimension centre subtracted from points and means before the products are formed (NULL = none; any value
+// gives the same mathematics, a centre near the data keeps the fp32 rounding small)
 cudaError_t launch_lse_fp32(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu,
-                            const float* w2, const double* c2d, double* logZ2, double* llpart);
+                            const float* w2, const double* c2d, const float* g, double* logZ2, double* llpart);
 cudaError_t launch_mstep_fp32(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu,
-                              const float* w2, const double* c2d, const double* logZ2, float* partials,
+                              const float* w2, const double* c2d, const float* g, const double* logZ2, float* partials,
                               const Fp32Plan& plan);
 // run_if: NULL, or a device flag: the kernel does nothing unless run_if[0] != 0.
 // gather: NULL, or device row indices: the points are X[gather[0 .. min(n, *gather_count))], and the outputs go to those
 // rows of idx / resp (n then bounds the number of gathered points, and sizes the grid).
 cudaError_t launch_topm_fp32(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu,
-                             const float* w2, const double* c2d, int m, int32_t* idx, float* resp,
+                             const float* w2, const double* c2d, const float* g, int m, int32_t* idx, float* resp,
                              const int* run_if = nullptr, const int32_t* gather = nullptr, const int* gather_count = nullptr);
 
 // ---- shared by all paths -------------------------------------------------------------------------------------

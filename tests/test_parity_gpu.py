@@ -450,6 +450,28 @@ def test_topm_exact_ties_go_to_the_smaller_index(fg, ctx):
     np.testing.assert_allclose(resp.cpu().numpy(), 1 / K, rtol=1e-5)
 
 
+def test_data_far_from_the_origin(fg, ctx):
+    """All points and means sit 300 standard deviations from the origin: the FP32 kernels form their products about the
+    centre of the means, so the offset costs no precision; the tensor path finds every component ill-conditioned for its
+    expanded form and recomputes what matters exactly."""
+    rng = np.random.default_rng(21)
+    N, D, K = 4000, 64, 96
+    X, pi, mu, var = _random_mixture(rng, N, D, K, spread=1.5)
+    X = (X + 300.0).astype(np.float32)
+    mu = (mu + 300.0).astype(np.float32)
+    s = data_scale(X)
+    ref = orc.em_step(X, pi, mu, var)
+    idx_r, resp_r, next_r = orc.topm(X, pi, mu, var, 3)
+    for path in _paths(fg, D, K):
+        ctx.gmm_set_path(path)
+        got = _gpu_step(ctx, _t(X), pi, mu, var)
+        assert abs(got[3] - ref[3]) <= 1e-5 * abs(ref[3]), path
+        assert_stats_close(N, s, got[:3], ref[:3], f"path {path}, data far from the origin")
+        idx_g, resp_g = ctx.gmm_assign_topm(_t(X), _t(pi), _t(mu), _t(var), 3)
+        torch.cuda.synchronize()
+        assert_topm_matches(idx_g.cpu().numpy(), resp_g.cpu().numpy(), idx_r, resp_r, next_r, what=f"path {path}, far from the origin")
+
+
 def test_scratch_does_not_grow_with_n(fg, ctx):
     assert fg.gmm_scratch_bytes(128, 1024) == fg.gmm_scratch_bytes(128, 1024)
     spec = synth.CONFIGS[2]

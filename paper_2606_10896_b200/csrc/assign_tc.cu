@@ -465,7 +465,8 @@ struct RefineArgs {
     const float* mu; const float* w2; const float* c2;
     int m; int32_t* idx_out; float* resp_out;
     float e_launch; int n_ill;
-    int32_t* unc_rows; int* unc_count;      // rows left to the exact kernel, and their number
+    int32_t* unc_rows; int* unc_count;      // rows left to the exact kernel (row + row_offset), and their number
+    int row_offset;                         // position of this piece inside the window of pieces that share the list
 };
 
 // One point, the whole warp: exact evaluation of what matters (see assign_refine_kernel).  Lane q < LIST holds the q-th
@@ -614,7 +615,7 @@ __device__ __forceinline__ void refine_point(const RefineArgs& g, const TcIllCac
     // Not certain (near ties, exact ties, too few finite candidates, broad posteriors): the point joins the list of rows
     // that the FP32 tile kernel evaluates against all K components afterwards.  (The order of the list varies from run to
     // run; the result of a row does not depend on it.)
-    if (lane == 0) g.unc_rows[atomicAdd(g.unc_count, 1)] = (int32_t)row;
+    if (lane == 0) g.unc_rows[atomicAdd(g.unc_count, 1)] = (int32_t)row + g.row_offset;
 }
 
 // A warp takes 32 consecutive points.  First every lane looks at one point on its own: it merges the records of the two
@@ -627,11 +628,11 @@ __global__ void __launch_bounds__(256)
 assign_refine_kernel(const float* __restrict__ rec, const float* __restrict__ X, int64_t n, int D, int K,
                      const float* __restrict__ mu, const float* __restrict__ w2, const float* __restrict__ c2,
                      const int* __restrict__ flags, const TcIllCache* __restrict__ ill_cache, int m, int32_t* __restrict__ idx_out,
-                     float* __restrict__ resp_out, int32_t* __restrict__ unc_rows, int* __restrict__ unc_count) {
+                     float* __restrict__ resp_out, int32_t* __restrict__ unc_rows, int* __restrict__ unc_count, int row_offset) {
     if (flags[3] != 0) return;
     constexpr int RECW = assign_recw(LIST);
     RefineArgs g;
-    g.unc_rows = unc_rows; g.unc_count = unc_count;
+    g.unc_rows = unc_rows; g.unc_count = unc_count; g.row_offset = row_offset;
     g.X = X; g.n = n; g.D = D; g.K = K; g.mu = mu; g.w2 = w2; g.c2 = c2; g.m = m; g.idx_out = idx_out; g.resp_out = resp_out;
     g.e_launch = __int_as_float(flags[1]);          // error bound of the approximate logits from the parameters
     g.n_ill = flags[2];                             // ill-conditioned components (<= TC_MAX_ILL): left out of the approximate pass
@@ -731,8 +732,8 @@ assign_refine_kernel(const float* __restrict__ rec, const float* __restrict__ X,
 
 template <int LIST>
 cudaError_t launch_assign_t(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu, const float* w2,
-                            const float* c2, const TcBuffers& tb, float* rec, int32_t* unc_rows, int* unc_count, int m, int32_t* idx,
-                            float* resp, int* status) {
+                            const float* c2, const TcBuffers& tb, float* rec, int32_t* unc_rows, int* unc_count, int row_offset, int m,
+                            int32_t* idx, float* resp, int* status) {
     const TcPlan pl = tc_plan(D, K, 148);
     AssignParams p;
     p.n = n; p.n_chunks = pl.CL; p.n_ks = pl.n_ks;
@@ -763,13 +764,11 @@ cudaError_t launch_assign_t(cudaStream_t s, const float* X, int64_t n, int D, in
     assign_tc_kernel<LIST><<<grid, AT_THREADS, ASM_BYTES, s>>>(p, tm_yhi, tm_ylo, tm_phi, tm_plo);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    e = cudaMemsetAsync(unc_count, 0, sizeof(int), s);
-    if (e != cudaSuccess) return e;
     const int64_t batches = (n + 31) / 32;                                         // a warp takes 32 points at a time
     const int64_t warps_wanted = batches < (int64_t)sms * 64 ? batches : (int64_t)sms * 64;
     const unsigned rgrid = (unsigned)((warps_wanted + 7) / 8);
     assign_refine_kernel<LIST, (LIST <= 6 ? 4 : GMM_MAX_TOPM)><<<rgrid, 256, 0, s>>>(rec, X, n, D, K, mu, w2, c2, tb.flags, tb.ill_cache, m, idx,
-                                                                               resp, unc_rows, unc_count);
+                                                                               resp, unc_rows, unc_count, row_offset);
     return cudaGetLastError();
 }
 
@@ -789,11 +788,11 @@ extern "C" void gmm_debug_refine_counts(unsigned long long* out) {
 size_t assign_tc_record_bytes(int m) { return (size_t)2 * assign_recw(m <= 4 ? 6 : 10) * sizeof(float); }
 
 cudaError_t launch_assign_tc(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu, const float* w2,
-                             const float* c2, const TcBuffers& tb, float* rec, int32_t* unc_rows, int* unc_count, int m, int32_t* idx,
-                             float* resp, int* status) {
+                             const float* c2, const TcBuffers& tb, float* rec, int32_t* unc_rows, int* unc_count, int row_offset, int m,
+                             int32_t* idx, float* resp, int* status) {
     if (n < 1 || n > TC_YPOINTS || m < 1 || m > GMM_MAX_TOPM) return cudaErrorInvalidValue;
-    if (m <= 4) return launch_assign_t<6>(s, X, n, D, K, mu, w2, c2, tb, rec, unc_rows, unc_count, m, idx, resp, status);
-    return launch_assign_t<10>(s, X, n, D, K, mu, w2, c2, tb, rec, unc_rows, unc_count, m, idx, resp, status);
+    if (m <= 4) return launch_assign_t<6>(s, X, n, D, K, mu, w2, c2, tb, rec, unc_rows, unc_count, row_offset, m, idx, resp, status);
+    return launch_assign_t<10>(s, X, n, D, K, mu, w2, c2, tb, rec, unc_rows, unc_count, row_offset, m, idx, resp, status);
 }
 
 }  // namespace fg

@@ -165,26 +165,17 @@ struct TopList {
 // M == 0: log-sum-exp only.  M > 0: also the top-M components per point.
 // ACC is the type the logits are carried in: float for D <= 128, double beyond (see tile_quadratic).  The exponentials
 // always take a float argument formed AFTER the subtraction of the reference, so large common offsets cancel exactly.
+// One tile of TP points (tile number blk) of the log-sum-exp / top-m pass: see lse_kernel.
 template <int M, typename ACC>
-__global__ void __launch_bounds__(NTHREADS)
-lse_kernel(const float* __restrict__ X, int64_t n, int D, int K, const float* __restrict__ mu,
-           const float* __restrict__ w2, const double* __restrict__ c2, const float* __restrict__ g,
-           double* __restrict__ logZ2, double* __restrict__ llpart, int m_out, int32_t* __restrict__ idx_out,
-           float* __restrict__ resp_out, const int* __restrict__ run_if, const int32_t* __restrict__ gather,
-           const int* __restrict__ gather_count) {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    // run_if: the launch does nothing unless run_if[0] != 0 (the tensor-core assignment covers the other case)
-    if (run_if && run_if[0] == 0) return;
-    // gather: the points are X[gather[0 .. *gather_count)] (top-m outputs go to those rows); CTAs beyond the count leave
-    if (gather) {
-        const int64_t cnt = *gather_count;
-        n = cnt < n ? cnt : n;
-        if ((int64_t)blockIdx.x * TP >= n) return;
-    }
+__device__ __forceinline__ void lse_tile(unsigned char* smem_raw, int64_t blk, const float* __restrict__ X, int64_t n, int D, int K,
+                                         const float* __restrict__ mu, const float* __restrict__ w2, const double* __restrict__ c2,
+                                         const float* __restrict__ g, double* __restrict__ logZ2, double* __restrict__ llpart,
+                                         int m_out, int32_t* __restrict__ idx_out, float* __restrict__ resp_out,
+                                         const int32_t* __restrict__ gather) {
     TileSmem& sm = *reinterpret_cast<TileSmem*>(smem_raw);
     __shared__ double ll_s[TP];
     const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
-    const int64_t row0 = (int64_t)blockIdx.x * TP;
+    const int64_t row0 = blk * TP;
     const ACC NEG_INF = (ACC)(-CUDART_INF_F);
 
     ACC m_run[4];
@@ -294,8 +285,32 @@ lse_kernel(const float* __restrict__ X, int64_t n, int D, int K, const float* __
         if (tid == 0) {
             double s = 0.0;
             for (int i = 0; i < TP; ++i) s += ll_s[i];
-            llpart[blockIdx.x] = s;
+            llpart[blk] = s;
         }
+    }
+}
+
+template <int M, typename ACC>
+__global__ void __launch_bounds__(NTHREADS)
+lse_kernel(const float* __restrict__ X, int64_t n, int D, int K, const float* __restrict__ mu,
+           const float* __restrict__ w2, const double* __restrict__ c2, const float* __restrict__ g,
+           double* __restrict__ logZ2, double* __restrict__ llpart, int m_out, int32_t* __restrict__ idx_out,
+           float* __restrict__ resp_out, const int* __restrict__ run_if, const int32_t* __restrict__ gather,
+           const int* __restrict__ gather_count) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    // run_if: the launch does nothing unless run_if[0] != 0 (the tensor-core assignment covers the other case)
+    if (run_if && run_if[0] == 0) return;
+    if (!gather) {                                   // one CTA per tile
+        lse_tile<M, ACC>(smem_raw, blockIdx.x, X, n, D, K, mu, w2, c2, g, logZ2, llpart, m_out, idx_out, resp_out, nullptr);
+        return;
+    }
+    // gather: the points are X[gather[0 .. *gather_count)] (top-m outputs go to those rows).  The count is only known on
+    // the device, so the grid is fixed and small and its CTAs stride over the tiles of the list.
+    const int64_t cnt = *gather_count;
+    n = cnt < n ? cnt : n;
+    for (int64_t blk = blockIdx.x; blk * TP < n; blk += gridDim.x) {
+        lse_tile<M, ACC>(smem_raw, blk, X, n, D, K, mu, w2, c2, g, logZ2, llpart, m_out, idx_out, resp_out, gather);
+        __syncthreads();                             // the next tile reuses the shared memory
     }
 }
 
@@ -660,7 +675,8 @@ static cudaError_t launch_topm_t(cudaStream_t s, const float* X, int64_t n, int 
     if (need > smem) smem = need;
     cudaError_t e = cudaFuncSetAttribute(lse_kernel<M, ACC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    const unsigned blocks = (unsigned)((n + TP - 1) / TP);
+    unsigned blocks = (unsigned)((n + TP - 1) / TP);
+    if (gather && blocks > 592) blocks = 592;          // the listed rows are few: at most 4 CTAs per SM stride over them
     lse_kernel<M, ACC><<<blocks, NTHREADS, smem, s>>>(X, n, D, K, mu, w2, c2d, g, nullptr, nullptr, m, idx, resp, run_if, gather, gather_count);
     return cudaGetLastError();
 }

@@ -79,11 +79,12 @@ cudaError_t tc_make_plane_map(CUtensorMap* tm, void* base, int64_t rows, int box
 // with ill_list = true.  Both kernels return at once when tb.flags[3] != 0 (more than TC_MAX_ILL ill-conditioned
 // components): the caller then runs the FP32 kernels, gated the other way.
 size_t assign_tc_record_bytes(int m);
-// unc_rows [n] / unc_count [1]: receive the rows whose result is not certain (not written to idx / resp): the caller runs
-// launch_topm_fp32 over them (gather mode).
+// unc_rows / unc_count [1]: the rows whose result is not certain (not written to idx / resp) are appended as row +
+// row_offset at position (*unc_count)++ (the caller zeroes the count and may let several pieces share one list): the
+// caller runs launch_topm_fp32 over them (gather mode).
 cudaError_t launch_assign_tc(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu, const float* w2,
-                             const float* c2, const TcBuffers& tb, float* rec, int32_t* unc_rows, int* unc_count, int m,
-                             int32_t* idx, float* resp, int* status);
+                             const float* c2, const TcBuffers& tb, float* rec, int32_t* unc_rows, int* unc_count, int row_offset,
+                             int m, int32_t* idx, float* resp, int* status);
 cudaError_t launch_reduce_tc(cudaStream_t s, int D, int K, int Q, const TcBuffers& tb, double* Nk, double* S1,
                              double* S2, bool accumulate);
 

@@ -666,22 +666,36 @@ int assign_topm_impl(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, cons
         KL(launch_ill_cache_tc(ctx->stream, D, mu, ctx->w2(), ctx->c2(), tb));
         const int64_t piece = ctx->tc_piece;
         const int64_t cap = N < piece ? N : piece;
+        constexpr int WINDOW = 8;            // pieces that share one list of uncertain rows (and one exact pass over it)
+        const int64_t win_cap = (N < WINDOW * piece) ? N : WINDOW * piece;
         const size_t rec_bytes = align256((size_t)cap * assign_tc_record_bytes(m));
-        const size_t need = rec_bytes + align256((size_t)cap * sizeof(int32_t)) + 256;       // records, uncertain rows, their count
+        const size_t need = rec_bytes + align256((size_t)win_cap * sizeof(int32_t)) + 256;   // records, uncertain rows, their count
         CHECK(grow_buffer(ctx, &ctx->at_scratch, &ctx->at_scratch_bytes, need, "the assignment records"));
         unsigned char* base = static_cast<unsigned char*>(ctx->at_scratch);
         int32_t* unc_rows = reinterpret_cast<int32_t*>(base + rec_bytes);
         int* unc_count = reinterpret_cast<int*>(base + need - 256);
+        int in_window = 0;
+        int64_t win_start = 0;
         for (int64_t off = 0; off < N; off += piece) {
             const int64_t cnt = (N - off < piece) ? (N - off) : piece;
+            if (in_window == 0) {
+                win_start = off;
+                CU(cudaMemsetAsync(unc_count, 0, sizeof(int), ctx->stream));
+            }
             CHECK(prof_begin(ctx));
             KL(launch_transform_tc(ctx->stream, X + off * D, cnt, D, tb));
             KL(launch_assign_tc(ctx->stream, X + off * D, cnt, D, K, mu, ctx->w2(), ctx->c2(), tb, reinterpret_cast<float*>(base),
-                                unc_rows, unc_count, m, idx + off * m, resp + off * m, &ctx->result()->status));
+                                unc_rows, unc_count, (int)(off - win_start), m, idx + off * m, resp + off * m, &ctx->result()->status));
             ctx->launches++;
-            // the rows the refinement was not certain about: all K components exactly, by the FP32 tile kernel
-            KL(launch_topm_fp32(ctx->stream, X + off * D, cnt, D, K, mu, ctx->w2(), ctx->c2d(), ctx->center(), m, idx + off * m, resp + off * m,
-                                nullptr, unc_rows, unc_count));
+            ++in_window;
+            if (in_window == WINDOW || off + piece >= N) {
+                // The rows the refinement was not certain about, of the whole window: all K components exactly, by the FP32
+                // tile kernel.  (One launch per window: with a few hundred rows per piece a launch per piece is all latency.)
+                const int64_t win_rows = off + cnt - win_start;
+                KL(launch_topm_fp32(ctx->stream, X + win_start * D, win_rows, D, K, mu, ctx->w2(), ctx->c2d(), ctx->center(), m,
+                                    idx + win_start * m, resp + win_start * m, nullptr, unc_rows, unc_count));
+                in_window = 0;
+            }
             CHECK(prof_end(ctx));
         }
         run_fp32_if = tb.flags + 3;

@@ -134,8 +134,8 @@ int gmm_fit(gmm_ctx* ctx, const float* X, int64_t N, int D, int K,
  * against all K components exactly; components whose responsibility for a point is below 4.8e-7 keep the order and
  * the values of the selection pass (inside the 1e-6 tie width).  Parameters with more than 256 ill-conditioned
  * components run on the FP32 kernels (decided on the device; gmm_last_path then still reports the tensor path).  The
- * first call allocates a buffer of 128 or 192 bytes (m <= 4, m > 4) per point of one piece of at most 2^19 points,
- * outside gmm_scratch_bytes. */
+ * first call allocates a work buffer outside gmm_scratch_bytes: 128 or 192 bytes (m <= 4, m > 4) per point of one piece
+ * of at most 2^19 points plus 4 bytes per point of eight pieces (84 MB or 118 MB at most, independent of N). */
 int gmm_assign_topm(gmm_ctx* ctx, const float* X, int64_t N, int D, int K,
                     const float* pi, const float* mu, const float* var, int m,
                     int32_t* idx, float* resp);

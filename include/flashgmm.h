@@ -64,7 +64,7 @@ int gmm_destroy(gmm_ctx* ctx);
 /* Select the kernel path for later calls (default GMM_PATH_AUTO).  GMM_EUNSUPPORTED is reported by the compute
  * call, not here, if a forced path cannot run the shape. */
 int gmm_set_path(gmm_ctx* ctx, int path);
-/* 1 if the tensor-core path can run shape (D, K) (D <= 128 and K <= 1024), else 0; GMM_PATH_AUTO uses it whenever
+/* 1 if the tensor-core path can run shape (D, K) (D <= 128 and K <= 4096), else 0; GMM_PATH_AUTO uses it whenever
  * this returns 1.  Components too ill-conditioned for the expanded quadratic form (sum_d mu^2 / var beyond what a
  * 22-bit split resolves, e.g. a component collapsed onto one point) have their competitive logits recomputed
  * exactly inside the kernel. */
@@ -127,8 +127,7 @@ int gmm_fit(gmm_ctx* ctx, const float* X, int64_t N, int D, int K,
  * clusters with the largest responsibilities, which the caller thresholds with tau = 1/K).
  *   idx [N x m] int32 and resp [N x m] float32, device outputs; per point descending by responsibility, ties to the
  *   smaller component index.  1 <= m <= min(K, GMM_MAX_TOPM).  Asynchronous on the stream.
- * Where the tensor-core path applies (the rule of gmm_em_step, and also K up to 4096 at D <= 128, which only the
- * assignment kernels take) the logits of all components come from the tensor cores
+ * Where the tensor-core path applies (the rule of gmm_em_step) the logits of all components come from the tensor cores
  * as a selection pass and the best few per point are recomputed exactly in fp32, so indices and values are those of the
  * FP32 kernels; a point whose selection is not certain within the error bound of the selection pass is evaluated
  * against all K components exactly; components whose responsibility for a point is below 4.8e-7 keep the order and

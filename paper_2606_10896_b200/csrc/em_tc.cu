@@ -135,6 +135,44 @@ __device__ __forceinline__ bool xslot_wait_all(const XSlot* q, int CL, uint32_t 
 }
 
 
+// Groups of more than 8 CTAs (K > 1024), used by the BIG instantiation of the kernel only (the common instantiation
+// contains none of this, so its register allocation is not touched).
+// The (max, sum) pairs of the CL source CTAs are collected 8 at a time and merged as they come: mi = max, Z = sum of
+// s 2^(m - mi).
+__device__ __forceinline__ bool xslot_collect_many(const XSlot* ring, int CL, uint32_t tag, float& mi_out, float& Z_out,
+                                                volatile int* abort_flag, int* status) {
+    float mi = -CUDART_INF_F, Z = 0.f;
+    bool all = true;
+    for (int cb = 0; cb < CL; cb += 8) {
+        float2 e[8];
+        const int nc = (CL - cb < 8) ? (CL - cb) : 8;
+        if (!xslot_wait_all(ring + cb * 64, nc, tag, e, abort_flag, status)) all = false;
+        float m8 = mi;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) m8 = fmaxf(m8, e[c].x);
+        const float m8_safe = (m8 == -CUDART_INF_F) ? 0.f : m8;
+        Z = (mi == -CUDART_INF_F) ? 0.f : Z * fast_ex2(mi - m8_safe);
+#pragma unroll
+        for (int c = 0; c < 8; ++c) Z += (e[c].x == -CUDART_INF_F) ? 0.f : e[c].y * fast_ex2(e[c].x - m8_safe);
+        mi = m8;
+    }
+    mi_out = mi;
+    Z_out = Z;
+    return all;
+}
+// The lower-bound slots beyond the first 32 of a point (slot s at q + 64 s): lane l takes slots 32 + l, 64 + l, ...; lb
+// becomes the maximum with what it already holds.  Returns false if a slot does not carry the tag yet.
+__device__ __forceinline__ bool xslot_more_bounds(const XSlot* q, int nslots, uint32_t tag, int lane, float& lb) {
+    bool ok = true;
+    for (int sb = 32 + lane; sb < nslots; sb += 32) {
+        uint32_t v[4];
+        xslot_load(q + sb * 64, v);
+        if (v[1] == tag && v[3] == tag) lb = fmaxf(lb, __uint_as_float(v[0]));
+        else ok = false;
+    }
+    return ok;
+}
+
 // ---- warp reduce-scatter butterflies over 64 per-thread values: afterwards lane l holds the reduction (over the
 //      32 lanes) for points 2l and 2l+1.  62 shuffles instead of 64 x 5.
 template <int HALF, bool IS_MAX>
@@ -198,6 +236,7 @@ struct TcKernelParams {
 #endif
 };
 
+template <bool BIG>      // BIG: groups of more than 8 CTAs (1024 < K <= 4096)
 __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams p, const __grid_constant__ CUtensorMap tm_hi,
                                                             const __grid_constant__ CUtensorMap tm_lo) {
     extern __shared__ unsigned char smem_raw[];
@@ -419,6 +458,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                                     if (v[1] == tag && v[3] == tag) lbv[b8] = __uint_as_float(v[0]);
                                     else ok = false;
                                 }
+                                if (BIG && jb[b8] >= 0) ok = xslot_more_bounds(ring + jb[b8], 4 * p.CL, tag, lane, lbv[b8]) && ok;
                             }
                             if (__all_sync(0xffffffffu, ok)) break;
                             bool give_up = *abort_flag != 0;
@@ -530,24 +570,30 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                 // (test hook: one CTA stays silent for the first tile, so that its peers' bounded waits run out)
                 if (!(p.test_silent_rank == (int)rank && cluster_id == 0 && i == 0)) xslot_write(ring + rank * 64, mc, sc, tag);
                 TOC(tk_, 3);
-                float2 e[8];
+                float mi = -CUDART_INF_F, mi_safe = 0.f, Z = 0.f;
+                if (!BIG) {
+                    float2 e[8];
 #ifdef FLASHGMM_DEBUG
-                if (p.order & 64) {           // what-if timing only (results are wrong): do not wait for the peers
+                    if (p.order & 64) {           // what-if timing only (results are wrong): do not wait for the peers
 #pragma unroll
-                    for (int c = 0; c < 8; ++c) e[c] = make_float2(mc, sc);
-                } else
+                        for (int c = 0; c < 8; ++c) e[c] = make_float2(mc, sc);
+                    } else
 #endif
-                if (!xslot_wait_all(ring, p.CL, tag, e, abort_flag, p.status)) alive = false;
-                float mi = -CUDART_INF_F;
+                    if (!xslot_wait_all(ring, p.CL, tag, e, abort_flag, p.status)) alive = false;
 #pragma unroll
-                for (int c = 0; c < 8; ++c) mi = fmaxf(mi, e[c].x);
-                TOC(tk_, 4);
-                if (gtid == 0) TRACE(2, i);
-                const float mi_safe = (mi == -CUDART_INF_F) ? 0.f : mi;
-                float Z = 0.f;
+                    for (int c = 0; c < 8; ++c) mi = fmaxf(mi, e[c].x);
+                    TOC(tk_, 4);
+                    if (gtid == 0) TRACE(2, i);
+                    mi_safe = (mi == -CUDART_INF_F) ? 0.f : mi;
 #pragma unroll
-                for (int c = 0; c < 8; ++c)
-                    Z += (e[c].x == -CUDART_INF_F) ? 0.f : e[c].y * fast_ex2(e[c].x - mi_safe);
+                    for (int c = 0; c < 8; ++c)
+                        Z += (e[c].x == -CUDART_INF_F) ? 0.f : e[c].y * fast_ex2(e[c].x - mi_safe);
+                } else {
+                    if (!xslot_collect_many(ring, p.CL, tag, mi, Z, abort_flag, p.status)) alive = false;
+                    TOC(tk_, 4);
+                    if (gtid == 0) TRACE(2, i);
+                    mi_safe = (mi == -CUDART_INF_F) ? 0.f : mi;
+                }
                 TOC(tk_, 19);
                 const bool valid = pt < nvalid;
                 const float inv = (valid && Z > 0.f) ? __fdividef(RSCALE, Z) : 0.f;
@@ -1233,7 +1279,7 @@ void tc_set_test_hooks(int silent_rank, unsigned long long wait_limit_ns) {
 }
 void tc_set_order(int o) { g_tc_order = o; }
 
-bool tc_supports(int D, int K) { return D >= 1 && D <= 128 && K >= 1 && K <= 1024; }
+bool tc_supports(int D, int K) { return D >= 1 && D <= 128 && K >= 1 && K <= TC_MAX_K; }
 // The assignment kernels walk over the components in chunks of 128 inside one CTA: no group of CTAs, so K may be larger.
 bool tc_assign_supports(int D, int K) { return D >= 1 && D <= 128 && K >= 1 && K <= TC_ASSIGN_MAX_K; }
 
@@ -1310,6 +1356,7 @@ cudaError_t tc_make_plane_map(CUtensorMap* tm, void* base, int64_t rows, int box
 cudaError_t launch_em_tc(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu, const float* w2,
                          const float* c2, const TcBuffers& tb, int Q, int flush_tiles, int* status) {
     const TcPlan pl = tc_plan(D, K, 148);
+    const bool big = pl.CL > 8;
     TcKernelParams p;
     p.X = X; p.n = n; p.D = D; p.K = K; p.CL = pl.CL; p.Q = Q; p.n_ks = pl.n_ks;
     p.flush = (flush_tiles < 2) ? 2 : (flush_tiles & ~1);
@@ -1331,7 +1378,7 @@ cudaError_t launch_em_tc(cudaStream_t s, const float* X, int64_t n, int D, int K
     p.dbg_clk = g_tc_clk;
     p.dbg_trace = g_tc_trace;
 #endif
-    cudaError_t e = cudaFuncSetAttribute(em_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(big ? em_tc_kernel<true> : em_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e != cudaSuccess) return e;
     // exchange slots carry the tile number as their tag: clear what the previous launch left behind
     const size_t xbytes = (size_t)Q * 4 * pl.CL * 64 * sizeof(XSlot);
@@ -1359,20 +1406,22 @@ cudaError_t launch_em_tc(cudaStream_t s, const float* X, int64_t n, int D, int K
     if (e != cudaSuccess) return e;
     e = tc_make_plane_map(&tm_lo, tb.y_lo, rows_padded, TC_BN, n_atoms);
     if (e != cudaSuccess) return e;
-    return cudaLaunchKernelEx(&cfg, em_tc_kernel, p, tm_hi, tm_lo);
+    return big ? cudaLaunchKernelEx(&cfg, em_tc_kernel<true>, p, tm_hi, tm_lo) : cudaLaunchKernelEx(&cfg, em_tc_kernel<false>, p, tm_hi, tm_lo);
 }
 
 // Number of groups (of ceil(K/128) CTAs, one CTA per SM) that can be resident at once: the persistent grid size.
 cudaError_t tc_max_clusters(int D, int K, int* out) {
     const TcPlan pl = tc_plan(D, K, 148);
-    cudaError_t e = cudaFuncSetAttribute(em_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    const bool big = pl.CL > 8;
+    cudaError_t e = cudaFuncSetAttribute(big ? em_tc_kernel<true> : em_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e != cudaSuccess) return e;
     int dev = 0, sms = 0, per_sm = 0;
     e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, em_tc_kernel, NTHREADS, SMEM_BYTES);
+    e = big ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, em_tc_kernel<true>, NTHREADS, SMEM_BYTES)
+            : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, em_tc_kernel<false>, NTHREADS, SMEM_BYTES);
     if (e != cudaSuccess) return e;
     *out = (sms * per_sm) / pl.CL;
     return cudaSuccess;

@@ -11,7 +11,8 @@ constexpr int TC_BN = 64;            // points per tile
 constexpr int TC_FLUSH = 64;         // tiles between flushes of the TMEM accumulators into float64 partials (even)
 constexpr float TC_RSCALE = 4096.f;  // responsibilities are scaled by this power of two before the fp16 split
 constexpr int TC_PCOLS = 258;        // columns of a partial row: 256 statistics columns + N_k of each softmax group
-constexpr int TC_ASSIGN_MAX_K = 4096;  // the tensor-core assignment takes up to this many components (the E+M tile kernel: 1024)
+constexpr int TC_MAX_K = 4096;         // the E+M tile kernel: a group of ceil(K / 128) <= 32 CTAs covers the components
+constexpr int TC_ASSIGN_MAX_K = 4096;  // the tensor-core assignment takes up to this many components
 constexpr int TC_MAX_ILL = 256;       // ill-conditioned components the tensor-core assignment evaluates exactly for every point
 constexpr int64_t TC_YPOINTS = 1 << 19;   // points per launch of the tile kernel: capacity of the fp16 planes of Y in scratch
 constexpr size_t TC_YPLANE_BYTES = (size_t)TC_YPOINTS * 512;   // one plane: 256 fp16 values per point

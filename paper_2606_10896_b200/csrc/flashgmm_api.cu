@@ -284,7 +284,7 @@ int prepare_and_choose(gmm_ctx* ctx, int64_t N, int D, int K, const float* pi, c
     const bool tc_ok = ctx->lay.tc && ctx->tc_Q >= 1;
     const bool tc_auto = tc_ok && gmm_auto_path(D, K) == GMM_PATH_TENSOR;
     if (ctx->path == GMM_PATH_TENSOR && !tc_ok)
-        return fail(ctx, GMM_EUNSUPPORTED, "the tensor-core path needs D <= 128 and K <= 1024 (got D=%d K=%d)", D, K);
+        return fail(ctx, GMM_EUNSUPPORTED, "the tensor-core path needs D <= 128 and K <= 4096 (got D=%d K=%d)", D, K);
     if (ctx->path == GMM_PATH_FP32 || !tc_ok || (ctx->path == GMM_PATH_AUTO && !tc_auto)) {
         *path = GMM_PATH_FP32;
         return GMM_OK;

@@ -116,6 +116,17 @@ def test_tensor_ill_conditioned_mode_under_both_issue_orders(fg, order, monkeypa
         _teacher_forced(fg, c, synth.sample_host(spec), spec, 3, paths=[fg.GMM_PATH_TENSOR])
 
 
+def test_tensor_path_with_groups_of_more_than_8_ctas(fg, ctx):
+    """K = 2048: a group of 16 CTAs covers the components of a tile, so the (max, sum) pairs and, in the ill-conditioned
+    mode, the lower bounds are collected in several rounds.  Teacher-forced over 3 iterations on N = 4000 points: from the
+    second iteration on most components have collapsed and the exact-recomputation protocol runs."""
+    import dataclasses
+
+    spec = dataclasses.replace(synth.CONFIGS[2].with_n(4000), K=2048)
+    X = synth.sample_host(spec)
+    _teacher_forced(fg, ctx, X, spec, 3, paths=[fg.GMM_PATH_TENSOR])
+
+
 def test_tensor_path_accumulates_over_pieces(fg, monkeypatch):
     # The tensor path converts X to its fp16 planes and launches the tile kernel once per piece of points (2^19 by
     # default).  With pieces of 1024 points a 3000-point problem takes three launches, the last one ragged (952 points,
@@ -168,7 +179,8 @@ def test_config2_free_running_30_iterations(fg, ctx):
 
 
 @pytest.mark.parametrize("N,D,K", [(1, 1, 1), (127, 16, 8), (129, 96, 129), (64, 100, 1), (1000, 3, 65),
-                                    (257, 128, 128), (333, 130, 70), (500, 100, 200), (300, 30, 64), (700, 9, 1000)])
+                                    (257, 128, 128), (333, 130, 70), (500, 100, 200), (300, 30, 64), (700, 9, 1000),
+                                    (1500, 128, 4096), (900, 64, 2048), (700, 100, 1500)])
 def test_odd_shapes_one_step(fg, ctx, N, D, K):
     rng = np.random.Generator(np.random.PCG64(N * 1000 + D * 10 + K))
     mu = rng.normal(0, 2, (K, D))

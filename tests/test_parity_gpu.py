@@ -243,6 +243,7 @@ def test_auto_path_choice(fg, ctx):
     assert fg.gmm_auto_path(128, 1024) == fg.GMM_PATH_TENSOR
     assert fg.gmm_auto_path(16, 8) == fg.GMM_PATH_FP32
     assert fg.gmm_auto_path(768, 4096) == fg.GMM_PATH_FP32 and not fg.tensor_path_supports(768, 4096)
+    assert fg.gmm_auto_path(128, 4096) == fg.GMM_PATH_TENSOR and fg.gmm_auto_path(128, 4097) == fg.GMM_PATH_FP32
     X = _t(np.random.default_rng(0).normal(size=(500, 16)).astype(np.float32))
     pi, mu, var = _t(np.full(8, 1 / 8)), _t(np.random.default_rng(1).normal(size=(8, 16))), _t(np.ones((8, 16)))
     ctx.gmm_em_step(X, pi, mu, var)

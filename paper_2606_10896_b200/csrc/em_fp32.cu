@@ -581,20 +581,20 @@ __global__ void prepare_fp32_kernel(int D, int K, const float* __restrict__ pi, 
 }
 
 // g[d] = mean over the components of mu[k][d]: the centre the tile routine subtracts from points and means.  A block takes
-// 32 dimensions; its 8 warps sum every 8th component in float64 and the 8 partial sums are added in a fixed order.  A
+// 32 dimensions; its 32 warps sum every 32nd component in float64 and the 32 partial sums are added in a fixed order.  A
 // non-finite mean (reported through the status word by prepare_fp32_kernel) gives centre 0.
-__global__ void __launch_bounds__(256) center_fp32_kernel(int D, int K, const float* __restrict__ mu, float* __restrict__ g) {
-    __shared__ double part[8][32];
+__global__ void __launch_bounds__(1024) center_fp32_kernel(int D, int K, const float* __restrict__ mu, float* __restrict__ g) {
+    __shared__ double part[32][33];
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const int d = blockIdx.x * 32 + lane;
     double s = 0.0;
     if (d < D)
-        for (int k = w; k < K; k += 8) s += (double)mu[(size_t)k * D + d];
+        for (int k = w; k < K; k += 32) s += (double)mu[(size_t)k * D + d];
     part[w][lane] = s;
     __syncthreads();
     if (w == 0 && d < D) {
         double t = 0.0;
-        for (int j = 0; j < 8; ++j) t += part[j][lane];
+        for (int j = 0; j < 32; ++j) t += part[j][lane];
         const float c = (float)(t / (double)K);
         g[d] = isfinite(c) ? c : 0.f;
     }
@@ -640,7 +640,7 @@ size_t fp32_partial_floats(int D, int K) {
 }
 
 cudaError_t launch_center_fp32(cudaStream_t s, int D, int K, const float* mu, float* g) {
-    center_fp32_kernel<<<(unsigned)((D + 31) / 32), 256, 0, s>>>(D, K, mu, g);
+    center_fp32_kernel<<<(unsigned)((D + 31) / 32), 1024, 0, s>>>(D, K, mu, g);
     return cudaGetLastError();
 }
 

@@ -208,6 +208,16 @@ __device__ __forceinline__ void warp_reduce_scatter32(const float (&v)[32], floa
 }
 
 
+// s_d x of point r (0..63) of the tile held in a Y stage (the two fp16 planes, 128-byte swizzle as TMA wrote them)
+__device__ __forceinline__ float y_scaled_x(const unsigned char* stage, int r, int d) {
+    const int cx = 16 * (d >> 3) + (d & 7);              // column of dimension d (k-step interleaved order)
+    const int atom = cx >> 6, cc = cx & 63;
+    const uint32_t off = (uint32_t)(atom * 8192 + r * 128 + ((((cc >> 3) ^ (r & 7)) << 4) | ((cc & 7) << 1)));
+    const __half hi = *reinterpret_cast<const __half*>(stage + off);
+    const __half lo = *reinterpret_cast<const __half*>(stage + SM_YLO + off);
+    return __half2float(hi) + __half2float(lo);
+}
+
 struct TcKernelParams {
     const float* X;
     int64_t n;
@@ -222,6 +232,9 @@ struct TcKernelParams {
     const float* mu;               // [K][D] means (exact recomputation)
     const float* w2;               // [K][D] (log2 e / 2) / var
     const float* c2;               // [K] log2 e (log pi - 1/2 sum log(2 pi var))
+    const int* dec_dim;            // [CL*128][8] ill-conditioned components: their 8 dimensions of largest weight (descending),
+    const float* dec_w;            // [CL*128][8] the weight there in units of the scaled data: (log2 e / 2) / (var s_d^2),
+    const float* dec_mu;           // [CL*128][8] and the scaled mean s_d mu
     double* partial;               // [Q][TC_PCOLS][CL*128]  (+=)
     double* llpart;                // [2 Q]
     XSlot* xg;                     // [Q][4][CL][64] exchange slots (zeroed before every launch)
@@ -236,7 +249,9 @@ struct TcKernelParams {
 #endif
 };
 
-template <bool BIG>      // BIG: groups of more than 8 CTAs (1024 < K <= 4096)
+// BIG: groups of more than 8 CTAs (1024 < K <= 4096).  TIGHT: the filter for launches in which many components are
+// ill-conditioned (see `tight` below); the host picks it from the count the previous preparation reported.
+template <bool BIG, bool TIGHT>
 __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams p, const __grid_constant__ CUtensorMap tm_hi,
                                                             const __grid_constant__ CUtensorMap tm_lo) {
     extern __shared__ unsigned char smem_raw[];
@@ -320,6 +335,11 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
         const float ck = p.ck[rank * 128 + kloc];
         const float illb = p.illb[rank * 128 + kloc];
         const bool any_ill = p.flags[0] != 0;
+        // Two filters for flagged components.  With few of them (large N / K: a few percent, truly collapsed ones) the test
+        // on the error bound alone discards nearly every pair, and anything more only adds instructions to every tile.
+        // With many (small N / K: half of the components narrow in a few dimensions) that test passes almost everything
+        // and the exact test on the decisive dimensions takes over (TIGHT; both give correct results on any input).
+        const bool tight = TIGHT && any_ill;
         float emax_w = illb;                                    // largest error bound among this warp's components
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) emax_w = fmaxf(emax_w, __shfl_xor_sync(0xffffffffu, emax_w, o));
@@ -393,14 +413,26 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
             // almost everything: a collapsed component is hopeless for every point but its own); the rare survivors
             // are checked against the group-wide bound read from the published slots and, if they pass, recomputed
             // exactly with direct differences in fp32, the whole warp working on one pair at a time.
-            // warp-level max per point (lane j ends up with point j)
-            warp_reduce_scatter32<true>(l, red, lane);
+            // warp-level max per point (lane j ends up with point j).  In a warp that has flagged components the maximum is
+            // taken over the well-conditioned ones only: that is a valid lower bound of the point's best log2 z (E = 0), a
+            // tight one, and it is also the maximum of everything that stays in play: a flagged pair either fails the
+            // tests below (its value lies 2^-40 below this bound or is removed) or is recomputed exactly, after which the
+            // maxima are formed again.
+            if (tight && emax_w > 0.f) {
+                float lt[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) lt[j] = (illb > 0.f) ? -CUDART_INF_F : l[j];
+                warp_reduce_scatter32<true>(lt, red, lane);
+            } else {
+                warp_reduce_scatter32<true>(l, red, lane);
+            }
             if (any_ill) {
                 // max_k (l_k - E_k) >= max_k l_k - max_k E_k: the warp maximum minus the warp's largest error bound is a
                 // valid lower bound (and for a warp without flagged lanes it is the maximum itself)
                 const uint32_t tag = (uint32_t)(i + 1);
                 XSlot* ring = xl + (size_t)(i & 3) * p.CL * 256 + p0;
-                const float lb_own = red - emax_w;                      // this warp's lower bound for point `lane`
+                // this warp's lower bound for point `lane`: see above, or max_k (l_k - E_k) >= max_k l_k - max_k E_k
+                const float lb_own = tight ? red : red - emax_w;
                 uint32_t mlo = 0;
                 if (emax_w > 0.f) {
 #ifdef FLASHGMM_DEBUG
@@ -409,11 +441,45 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
 #endif
                     // Local filter, by shuffles (no shared memory, no warp barrier: a barrier here would also wait for
                     // global stores in flight): bit j of mlo = point j of this lane's component may matter.
-                    const float reach = (illb > 0.f) ? illb + ILL_MARGIN : -CUDART_INF_F;
+                    // (only flagged lanes: in the tight mode a warp without a well-conditioned component has the bound -inf,
+                    // which every value reaches, also the -inf of a padded component)
+                    const bool flagged = illb > 0.f;
+                    const float reach = illb + ILL_MARGIN;
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
                         const float lbj = __shfl_sync(0xffffffffu, lb_own, j);
-                        if (j < nvalid && l[j] + reach >= lbj) mlo |= 1u << j;
+                        if (flagged && j < nvalid && l[j] + reach >= lbj) mlo |= 1u << j;
+                    }
+                    // For a component that is narrow in a few dimensions only, E is in the thousands and almost every pair
+                    // passes that test.  Such pairs are then tested exactly: c_k minus the terms of the component's 8
+                    // dimensions of largest weight is an upper bound of its log2 z, whatever the other dimensions add.  The
+                    // warp takes one flagged component at a time, lane j testing point j; the coordinates are read from
+                    // the tile's fp16 planes in shared memory.
+                    unsigned fl = tight ? __ballot_sync(0xffffffffu, mlo != 0u) : 0u;
+                    if (fl) {
+                        // (the planes were written by TMA: observing the stage's barrier makes them visible to these loads)
+                        bar_wait(BAR(B_YFULL0 + s), ph, abort_flag, p.status, false);
+                        const unsigned char* ystage = smem + SM_Y + s * SM_YSTAGE;
+                        while (fl) {
+                            const int f = __ffs(fl) - 1;
+                            fl &= fl - 1;
+                            const int kf = (int)rank * 128 + wq * 32 + f;
+                            const unsigned maskf = __shfl_sync(0xffffffffu, mlo, f);
+                            float ub = __ldg(p.c2 + kf);
+#pragma unroll
+                            for (int q8 = 0; q8 < 8; ++q8) {
+                                const int d = __ldg(p.dec_dim + kf * 8 + q8);
+                                const float x = y_scaled_x(ystage, p0 + lane, d);
+                                // (coordinates are clamped to +-240 when the planes are built: such a one proves nothing)
+                                const float w = (fabsf(x) < 239.f) ? __ldg(p.dec_w + kf * 8 + q8) : 0.f;
+                                const float diff = x - __ldg(p.dec_mu + kf * 8 + q8);
+                                ub -= w * diff * diff;
+                            }
+                            // 8: rounding of the 22-bit coordinates
+                            const bool keep = ((maskf >> lane) & 1u) && !(ub < lb_own - ILL_MARGIN - 8.f);
+                            const unsigned km = __ballot_sync(0xffffffffu, keep);
+                            if (lane == f) mlo = km;
+                        }
                     }
                 }
                 // publish AFTER the filter: peers read these slots only for the rare pairs that survive their own filter,
@@ -423,6 +489,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                 if (emax_w > 0.f) {
                     const int kglob = (int)rank * 128 + kloc;
                     bool fixed_any = false;
+                    uint32_t exact_mask = 0;                                 // points of this lane's component recomputed exactly
                     TOC(tk_, 29);
                     // Second filter, against the GROUP-wide lower bound of each point (the maximum of the bounds that all
                     // 4 CL warps of the group published).  That bound depends on the point only, so it is fetched once per
@@ -520,8 +587,17 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                             for (int jj = 0; jj < 32; ++jj)
                                 if (jj == j) l[jj] = val;
                             mlo &= ~(1u << j);
+                            exact_mask |= 1u << j;
                         }
                         fixed_any = true;
+                    }
+                    // Tight mode: the approximate value of a flagged component is never used: a pair that was not recomputed has been
+                    // shown to lie 2^-40 below the point's best value (and its approximation may be off by thousands, in
+                    // either direction), so it takes no further part.
+                    if (tight && illb > 0.f) {
+#pragma unroll
+                        for (int jj = 0; jj < 32; ++jj)
+                            if (!((exact_mask >> jj) & 1u)) l[jj] = -CUDART_INF_F;
                     }
                     __syncwarp();
                     TOC(tk_, 30);
@@ -1145,6 +1221,7 @@ __global__ void __launch_bounds__(128) tc_prepare_kernel(int D, int K, const flo
         if (k < K && cond > (double)cond_limit) {
             margin = (float)fmin(8.0 * cond, 1e30);       // E_k: error bound of the approximate log2 z (8 x the estimate)
             atomicOr(flags, 1);
+            atomicAdd(flags + 4, 1);                      // how many: the tile kernel picks its filter by their share
         }
         illb[k] = margin;
         // For the assignment kernels: an ill-conditioned component takes no part in the approximate selection (constant
@@ -1154,6 +1231,52 @@ __global__ void __launch_bounds__(128) tc_prepare_kernel(int D, int K, const flo
         if (k < K && margin == 0.f) {
             const float eb = (float)fmin(8.0 * cond, 1e30);
             if (eb > 0.f) atomicMax(flags + 1, __float_as_int(eb));
+        }
+    }
+}
+
+// One warp per ill-conditioned component (illb > 0): its 8 dimensions of largest weight, in descending order of the weight,
+// in units of the scaled data (the tile kernel reads s_d x from the fp16 planes): weight (log2 e / 2) / (var s_d^2), mean
+// s_d mu.  The tile kernel uses them for an exact upper bound of log2 z that costs a few shared-memory reads.
+__global__ void __launch_bounds__(256) tc_decisive_kernel(int D, int K, const float* __restrict__ mu, const float* __restrict__ var,
+                                                          const float* __restrict__ sd, const float* __restrict__ illb,
+                                                          int* __restrict__ dec_dim, float* __restrict__ dec_w,
+                                                          float* __restrict__ dec_mu) {
+    const int k = (int)((blockIdx.x * blockDim.x + threadIdx.x) >> 5), lane = threadIdx.x & 31;
+    if (k >= K || !(illb[k] > 0.f)) return;          // warp-uniform
+    float wv[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const int d = lane + 32 * j;
+        wv[j] = -1.f;
+        if (d < D) {
+            const float sdd = sd[d];
+            wv[j] = (0.72134752044448170368f / var[(size_t)k * D + d]) / (sdd * sdd);
+            if (!(wv[j] >= 0.f) || !isfinite(wv[j])) wv[j] = 0.f;
+        }
+    }
+    for (int r = 0; r < 8; ++r) {
+        float bv = wv[0];
+        int bd = lane;
+#pragma unroll
+        for (int j = 1; j < 4; ++j)
+            if (wv[j] > bv) { bv = wv[j]; bd = lane + 32 * j; }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+            const int od = __shfl_xor_sync(0xffffffffu, bd, o);
+            if (ov > bv || (ov == bv && od < bd)) { bv = ov; bd = od; }
+        }
+        if ((bd & 31) == lane) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (lane + 32 * j == bd) wv[j] = -1.f;          // taken
+        }
+        if (lane == 0) {
+            const bool have = bv >= 0.f;
+            dec_dim[k * 8 + r] = have ? bd : 0;
+            dec_w[k * 8 + r] = have ? bv : 0.f;
+            dec_mu[k * 8 + r] = have ? sd[bd] * mu[(size_t)k * D + bd] : 0.f;
         }
     }
 }
@@ -1297,7 +1420,7 @@ cudaError_t launch_prepare_tc(cudaStream_t s, int D, int K, const float* pi, con
                               const TcBuffers& tb, float cond_limit, int* status, bool ill_list) {
     const TcPlan pl = tc_plan(D, K, 148);
     (void)status;
-    cudaError_t e0 = cudaMemsetAsync(tb.flags, 0, 4 * sizeof(int), s);
+    cudaError_t e0 = cudaMemsetAsync(tb.flags, 0, 8 * sizeof(int), s);
     if (e0 != cudaSuccess) return e0;
     tc_scale_kernel<<<128, 128, 0, s>>>(D, K, pi, mu, var, tb.sd, tb.kap);
     cudaError_t e = cudaGetLastError();
@@ -1305,6 +1428,9 @@ cudaError_t launch_prepare_tc(cudaStream_t s, int D, int K, const float* pi, con
     tc_prepare_kernel<<<pl.Kpad, 128, 0, s>>>(D, K, pi, mu, var, tb.sd, tb.kap, tb.phi_img, tb.plo_img, tb.tk, tb.ck, tb.illb, cond_limit, tb.flags,
                                                   reinterpret_cast<uint32_t*>(tb.p_hi_rm), reinterpret_cast<uint32_t*>(tb.p_lo_rm),
                                                   reinterpret_cast<float2*>(tb.tkck));
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    tc_decisive_kernel<<<(unsigned)((K + 7) / 8), 256, 0, s>>>(D, K, mu, var, tb.sd, tb.illb, tb.dec_dim, tb.dec_w, tb.dec_mu);
     e = cudaGetLastError();
     if (e != cudaSuccess || !ill_list) return e;
     tc_ill_list_kernel<<<1, 1024, 0, s>>>(pl.Kpad, tb.illb, tb.ill_list, tb.flags);
@@ -1353,8 +1479,17 @@ cudaError_t tc_make_plane_map(CUtensorMap* tm, void* base, int64_t rows, int box
     return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
+namespace {
+cudaError_t set_smem_attr(bool big, bool tight) {
+    if (big) return tight ? cudaFuncSetAttribute(em_tc_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES)
+                          : cudaFuncSetAttribute(em_tc_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    return tight ? cudaFuncSetAttribute(em_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES)
+                 : cudaFuncSetAttribute(em_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+}
+}  // namespace
+
 cudaError_t launch_em_tc(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu, const float* w2,
-                         const float* c2, const TcBuffers& tb, int Q, int flush_tiles, int* status) {
+                         const float* c2, const TcBuffers& tb, int Q, int flush_tiles, bool tight, int* status) {
     const TcPlan pl = tc_plan(D, K, 148);
     const bool big = pl.CL > 8;
     TcKernelParams p;
@@ -1370,6 +1505,7 @@ cudaError_t launch_em_tc(cudaStream_t s, const float* X, int64_t n, int D, int K
     }
     p.phi_img = tb.phi_img; p.plo_img = tb.plo_img; p.tk = tb.tk; p.ck = tb.ck;
     p.illb = tb.illb; p.flags = tb.flags; p.mu = mu; p.w2 = w2; p.c2 = c2;
+    p.dec_dim = tb.dec_dim; p.dec_w = tb.dec_w; p.dec_mu = tb.dec_mu;
     p.partial = tb.partial; p.llpart = tb.llpart; p.status = status;
     p.xg = static_cast<XSlot*>(tb.xg); p.xl = static_cast<XSlot*>(tb.xl);
 #ifdef FLASHGMM_DEBUG
@@ -1378,7 +1514,7 @@ cudaError_t launch_em_tc(cudaStream_t s, const float* X, int64_t n, int D, int K
     p.dbg_clk = g_tc_clk;
     p.dbg_trace = g_tc_trace;
 #endif
-    cudaError_t e = cudaFuncSetAttribute(big ? em_tc_kernel<true> : em_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    cudaError_t e = set_smem_attr(big, tight);
     if (e != cudaSuccess) return e;
     // exchange slots carry the tile number as their tag: clear what the previous launch left behind
     const size_t xbytes = (size_t)Q * 4 * pl.CL * 64 * sizeof(XSlot);
@@ -1406,22 +1542,24 @@ cudaError_t launch_em_tc(cudaStream_t s, const float* X, int64_t n, int D, int K
     if (e != cudaSuccess) return e;
     e = tc_make_plane_map(&tm_lo, tb.y_lo, rows_padded, TC_BN, n_atoms);
     if (e != cudaSuccess) return e;
-    return big ? cudaLaunchKernelEx(&cfg, em_tc_kernel<true>, p, tm_hi, tm_lo) : cudaLaunchKernelEx(&cfg, em_tc_kernel<false>, p, tm_hi, tm_lo);
+    if (big) return tight ? cudaLaunchKernelEx(&cfg, em_tc_kernel<true, true>, p, tm_hi, tm_lo) : cudaLaunchKernelEx(&cfg, em_tc_kernel<true, false>, p, tm_hi, tm_lo);
+    return tight ? cudaLaunchKernelEx(&cfg, em_tc_kernel<false, true>, p, tm_hi, tm_lo) : cudaLaunchKernelEx(&cfg, em_tc_kernel<false, false>, p, tm_hi, tm_lo);
 }
 
 // Number of groups (of ceil(K/128) CTAs, one CTA per SM) that can be resident at once: the persistent grid size.
 cudaError_t tc_max_clusters(int D, int K, int* out) {
     const TcPlan pl = tc_plan(D, K, 148);
     const bool big = pl.CL > 8;
-    cudaError_t e = cudaFuncSetAttribute(big ? em_tc_kernel<true> : em_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    cudaError_t e = set_smem_attr(big, true);
     if (e != cudaSuccess) return e;
     int dev = 0, sms = 0, per_sm = 0;
     e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
-    e = big ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, em_tc_kernel<true>, NTHREADS, SMEM_BYTES)
-            : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, em_tc_kernel<false>, NTHREADS, SMEM_BYTES);
+    // (the same for every instantiation: one CTA per SM, by shared memory)
+    e = big ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, em_tc_kernel<true, true>, NTHREADS, SMEM_BYTES)
+            : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, em_tc_kernel<false, true>, NTHREADS, SMEM_BYTES);
     if (e != cudaSuccess) return e;
     *out = (sms * per_sm) / pl.CL;
     return cudaSuccess;

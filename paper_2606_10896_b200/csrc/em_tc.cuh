@@ -52,6 +52,9 @@ struct TcBuffers {
     float* tkck;              // [Kpad] pairs (t_k, c_k); c_k = -inf for ill-conditioned components
     int* ill_list;            // [Kpad] ascending indices of the ill-conditioned components (flags[2] of them)
     TcIllCache* ill_cache;    // filled by launch_ill_cache_tc
+    int* dec_dim;             // [Kpad][8] per ill-conditioned component: its 8 dimensions of largest weight,
+    float* dec_w;             // [Kpad][8] the weights there (units of the scaled data)
+    float* dec_mu;            // [Kpad][8] and the scaled means
 };
 
 bool tc_supports(int D, int K);          // the E+M tile kernel
@@ -67,9 +70,10 @@ cudaError_t launch_prepare_tc(cudaStream_t s, int D, int K, const float* pi, con
 // One pass over at most TC_YPOINTS points: X -> the two fp16 planes of Y in scratch (read by the tile kernel through TMA).
 cudaError_t launch_transform_tc(cudaStream_t s, const float* X, int64_t n, int D, const TcBuffers& tb);
 // n <= TC_YPOINTS points whose planes launch_transform_tc has written.
-// mu, w2, c2: the FP32 path's derived parameters (launch_prepare_fp32), used to recompute ill-conditioned logits exactly
+// mu, w2, c2: the FP32 path's derived parameters (launch_prepare_fp32), used to recompute ill-conditioned logits exactly.
+// tight: use the filter meant for launches in which many components are ill-conditioned (tb.flags[4] counts them).
 cudaError_t launch_em_tc(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu, const float* w2,
-                         const float* c2, const TcBuffers& tb, int Q, int flush_tiles, int* status);
+                         const float* c2, const TcBuffers& tb, int Q, int flush_tiles, bool tight, int* status);
 // After launch_prepare_tc(..., ill_list = true): fills tb.ill_cache for the first min(flags[2], TC_MAX_ILL) listed components.
 // w2, c2: the FP32 path's derived parameters (launch_prepare_fp32).
 cudaError_t launch_ill_cache_tc(cudaStream_t s, int D, const float* mu, const float* w2, const float* c2, const TcBuffers& tb);

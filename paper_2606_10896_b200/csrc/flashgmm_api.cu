@@ -18,7 +18,7 @@ namespace {
 struct DevResult {
     double ll[LL_SLOTS];
     int status;
-    int pad;
+    int n_ill;      // ill-conditioned components found by the tensor path's last preparation
 };
 
 constexpr size_t STAGE_BYTES = (size_t)128 << 20;   // per staging buffer of the host-streaming path
@@ -28,7 +28,7 @@ inline size_t align256(size_t b) { return (b + 255) & ~(size_t)255; }
 
 struct ScratchLayout {
     size_t w2, c2, c2d, center, partials, logZ2, llpart, result, stats, total;
-    size_t tc_phi, tc_plo, tc_tk, tc_ck, tc_sd, tc_kap, tc_illb, tc_flags, tc_xg, tc_xl, tc_partial, tc_llpart, tc_partial_bytes, tc_yhi, tc_ylo, tc_phirm, tc_plorm, tc_tkck, tc_illlist, tc_illcache;
+    size_t tc_phi, tc_plo, tc_tk, tc_ck, tc_sd, tc_kap, tc_illb, tc_flags, tc_xg, tc_xl, tc_partial, tc_llpart, tc_partial_bytes, tc_yhi, tc_ylo, tc_phirm, tc_plorm, tc_tkck, tc_illlist, tc_illcache, tc_decdim, tc_decw, tc_decmu;
     bool tc;
 };
 
@@ -48,7 +48,7 @@ ScratchLayout scratch_layout(int D, int K, bool planes) {
     L.result = take(sizeof(DevResult));
     L.stats = take(((size_t)K + 2 * KD) * 8);
     L.tc = tc_assign_supports(D, K);           // the assignment kernels' shapes include the E+M tile kernel's
-    L.tc_phi = L.tc_plo = L.tc_tk = L.tc_ck = L.tc_sd = L.tc_kap = L.tc_illb = L.tc_flags = L.tc_xg = L.tc_xl = L.tc_partial = L.tc_llpart = L.tc_yhi = L.tc_ylo = L.tc_phirm = L.tc_plorm = L.tc_tkck = L.tc_illlist = L.tc_illcache = 0;
+    L.tc_phi = L.tc_plo = L.tc_tk = L.tc_ck = L.tc_sd = L.tc_kap = L.tc_illb = L.tc_flags = L.tc_xg = L.tc_xl = L.tc_partial = L.tc_llpart = L.tc_yhi = L.tc_ylo = L.tc_phirm = L.tc_plorm = L.tc_tkck = L.tc_illlist = L.tc_illcache = L.tc_decdim = L.tc_decw = L.tc_decmu = 0;
     L.tc_partial_bytes = 0;
     if (L.tc) {
         const TcPlan pl = tc_plan(D, K, 160);       // an upper bound on the number of clusters
@@ -59,7 +59,7 @@ ScratchLayout scratch_layout(int D, int K, bool planes) {
         L.tc_sd = take(128 * 4);
         L.tc_kap = take(128 * 4);
         L.tc_illb = take((size_t)pl.Kpad * 4);
-        L.tc_flags = take(16);
+        L.tc_flags = take(32);
         if (tc_supports(D, K)) {                // what only the E+M tile kernel needs
             L.tc_xg = take((size_t)pl.Q * 4 * pl.CL * 64 * 16);
             L.tc_xl = take((size_t)pl.Q * 4 * pl.CL * 256 * 16);
@@ -72,6 +72,9 @@ ScratchLayout scratch_layout(int D, int K, bool planes) {
         L.tc_tkck = take((size_t)pl.Kpad * 8);
         L.tc_illlist = take((size_t)pl.Kpad * 4);
         L.tc_illcache = take(sizeof(TcIllCache));
+        L.tc_decdim = take((size_t)pl.Kpad * 8 * 4);
+        L.tc_decw = take((size_t)pl.Kpad * 8 * 4);
+        L.tc_decmu = take((size_t)pl.Kpad * 8 * 4);
     }
     if (L.tc && planes) {
         L.tc_yhi = take(TC_YPLANE_BYTES);
@@ -108,6 +111,7 @@ struct gmm_ctx {
     float tc_cond_scale = 1.5e-4f;
     int tc_flush = TC_FLUSH;
     int64_t tc_piece = TC_YPOINTS;   // points per launch of the tile kernel (<= capacity of the Y planes)
+    int tc_n_ill = 0;                // ill-conditioned components at the last result that was read back (picks the filter)
     // host-streaming path
     cudaStream_t copy_stream = nullptr;
     float* xstage[2] = {nullptr, nullptr};
@@ -154,6 +158,9 @@ struct gmm_ctx {
         b.tkck = reinterpret_cast<float*>(scratch + lay.tc_tkck);
         b.ill_list = reinterpret_cast<int*>(scratch + lay.tc_illlist);
         b.ill_cache = reinterpret_cast<TcIllCache*>(scratch + lay.tc_illcache);
+        b.dec_dim = reinterpret_cast<int*>(scratch + lay.tc_decdim);
+        b.dec_w = reinterpret_cast<float*>(scratch + lay.tc_decw);
+        b.dec_mu = reinterpret_cast<float*>(scratch + lay.tc_decmu);
         return b;
     }
 };
@@ -295,7 +302,9 @@ int prepare_and_choose(gmm_ctx* ctx, int64_t N, int D, int K, const float* pi, c
     float limit = ctx->tc_cond_limit;
     if (limit < 0.f) limit = ctx->tc_cond_scale * std::sqrt((float)((double)N / (double)K));
     KL(launch_prepare_tc(ctx->stream, D, K, pi, mu, var, ctx->tc(), limit, &ctx->result()->status));
-    ctx->launches++;   // launch_prepare_tc enqueues two kernels
+    ctx->launches += 2;   // launch_prepare_tc enqueues three kernels
+    // the number of ill-conditioned components travels back with the result: the next step picks its filter by it
+    CU(cudaMemcpyAsync(&ctx->result()->n_ill, ctx->tc().flags + 4, sizeof(int), cudaMemcpyDeviceToDevice, ctx->stream));
     *path = GMM_PATH_TENSOR;
     return GMM_OK;
 }
@@ -307,6 +316,12 @@ int accumulate_points(gmm_ctx* ctx, int path, const float* X, int64_t n, int D, 
         const TcBuffers tb = ctx->tc();
         const TcPlan pl = tc_plan(D, K, 160);
         const int Q = ctx->tc_Q;
+        // Which filter the tile kernel applies to ill-conditioned components (both are correct on any input).  With few
+        // points per component the flagged components are mostly narrow in a few dimensions, the test on their error
+        // bound passes nearly every pair and the exact test on their decisive dimensions pays; with many points per
+        // component they are collapsed singletons that the error-bound test already discards.  Decided from the count of
+        // the last preparation whose result was read back (none yet: the plain filter).
+        const bool tight = ctx->tc_n_ill > 0 && (n < (int64_t)512 * K || (int64_t)ctx->tc_n_ill * 8 > K);
         CU(cudaMemsetAsync(tb.partial, 0, (size_t)Q * pl.Kpad * TC_PCOLS * 8, ctx->stream));
         CU(cudaMemsetAsync(tb.llpart, 0, (size_t)Q * 16, ctx->stream));
         // The fp16 planes of Y are built once per launch-sized piece of X (not once per CTA of a group), so the tile kernel
@@ -316,7 +331,7 @@ int accumulate_points(gmm_ctx* ctx, int path, const float* X, int64_t n, int D, 
             const float* Xs = X + off * D;
             CHECK(prof_begin(ctx));
             KL(launch_transform_tc(ctx->stream, Xs, cnt, D, tb));
-            KL(launch_em_tc(ctx->stream, Xs, cnt, D, K, mu, ctx->w2(), ctx->c2(), tb, Q, ctx->tc_flush, &ctx->result()->status));
+            KL(launch_em_tc(ctx->stream, Xs, cnt, D, K, mu, ctx->w2(), ctx->c2(), tb, Q, ctx->tc_flush, tight, &ctx->result()->status));
             CHECK(prof_end(ctx));
         }
         KL(launch_reduce_ll(ctx->stream, tb.llpart, 2 * Q, &ctx->result()->ll[slot], true));
@@ -355,6 +370,7 @@ int read_result(gmm_ctx* ctx, int slot, double* loglik) {
     if (r.status & ST_BAD_VAR) return fail(ctx, GMM_ENUMERIC, "var must be finite and > 0");
     if (r.status & ST_BAD_PI) return fail(ctx, GMM_ENUMERIC, "pi must be finite and >= 0");
     if (r.status & ST_NONFINITE) return fail(ctx, GMM_ENUMERIC, "non-finite parameter");
+    ctx->tc_n_ill = r.n_ill;
     *loglik = r.ll[slot];
     if (!std::isfinite(*loglik)) return fail(ctx, GMM_ENUMERIC, "log-likelihood is not finite (%g)", *loglik);
     return GMM_OK;
@@ -662,7 +678,7 @@ int assign_topm_impl(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, cons
         const TcBuffers tb = ctx->tc();
         const float limit = ctx->tc_cond_limit >= 0.f ? ctx->tc_cond_limit : 0.01f;
         KL(launch_prepare_tc(ctx->stream, D, K, pi, mu, var, tb, limit, &ctx->result()->status, true));
-        ctx->launches += 2;
+        ctx->launches += 3;
         KL(launch_ill_cache_tc(ctx->stream, D, mu, ctx->w2(), ctx->c2(), tb));
         const int64_t piece = ctx->tc_piece;
         const int64_t cap = N < piece ? N : piece;

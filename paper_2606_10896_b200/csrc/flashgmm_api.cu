@@ -112,6 +112,7 @@ struct gmm_ctx {
     int tc_flush = TC_FLUSH;
     int64_t tc_piece = TC_YPOINTS;   // points per launch of the tile kernel (<= capacity of the Y planes)
     int tc_n_ill = 0;                // ill-conditioned components at the last result that was read back (picks the filter)
+    int tc_force_filter = -1;        // GMM_TC_FILTER=plain / tight: 0 / 1 (tests); -1: automatic
     // host-streaming path
     cudaStream_t copy_stream = nullptr;
     float* xstage[2] = {nullptr, nullptr};
@@ -321,7 +322,8 @@ int accumulate_points(gmm_ctx* ctx, int path, const float* X, int64_t n, int D, 
         // bound passes nearly every pair and the exact test on their decisive dimensions pays; with many points per
         // component they are collapsed singletons that the error-bound test already discards.  Decided from the count of
         // the last preparation whose result was read back (none yet: the plain filter).
-        const bool tight = ctx->tc_n_ill > 0 && (n < (int64_t)512 * K || (int64_t)ctx->tc_n_ill * 8 > K);
+        bool tight = ctx->tc_n_ill > 0 && (n < (int64_t)512 * K || (int64_t)ctx->tc_n_ill * 8 > K);
+        if (ctx->tc_force_filter >= 0) tight = ctx->tc_force_filter == 1;
         CU(cudaMemsetAsync(tb.partial, 0, (size_t)Q * pl.Kpad * TC_PCOLS * 8, ctx->stream));
         CU(cudaMemsetAsync(tb.llpart, 0, (size_t)Q * 16, ctx->stream));
         // The fp16 planes of Y are built once per launch-sized piece of X (not once per CTA of a group), so the tile kernel
@@ -405,6 +407,7 @@ int gmm_create(gmm_ctx** out, int device, void* cuda_stream) {
     ctx->device = device;
     ctx->stream = static_cast<cudaStream_t>(cuda_stream);
     if (const char* e = std::getenv("GMM_TC_COND_LIMIT")) ctx->tc_cond_limit = (float)std::atof(e);
+    if (const char* e = std::getenv("GMM_TC_FILTER")) ctx->tc_force_filter = (e[0] == 't') ? 1 : (e[0] == 'p' ? 0 : -1);
     if (const char* e = std::getenv("GMM_TC_FLUSH")) ctx->tc_flush = std::atoi(e);
     if (const char* e = std::getenv("GMM_TC_PIECE")) {
         const long long v = std::atoll(e);

@@ -104,6 +104,17 @@ def test_config2_cut_teacher_forced(fg, ctx):
     _teacher_forced(fg, ctx, synth.sample_host(spec), spec, 3)
 
 
+@pytest.mark.parametrize("filt", ["plain", "tight"])
+def test_tensor_ill_conditioned_mode_with_either_filter(fg, filt, monkeypatch):
+    # The tile kernel has two filters for the pairs of flagged components (the host picks one per launch from the number of
+    # points per component); either must give the right statistics on any input.  N = 3000 < 3 K: from the second
+    # iteration on most components are flagged.
+    monkeypatch.setenv("GMM_TC_FILTER", filt)
+    spec = synth.CONFIGS[2].with_n(3000)
+    with fg.Context(0) as c:
+        _teacher_forced(fg, c, synth.sample_host(spec), spec, 4, paths=[fg.GMM_PATH_TENSOR])
+
+
 @pytest.mark.parametrize("order", ["0", "1", "2"])
 def test_tensor_ill_conditioned_mode_under_both_issue_orders(fg, order, monkeypatch):
     # From the second iteration on, N=3000 < 3K leaves most components collapsed onto single points at the variance

@@ -496,6 +496,24 @@ def test_data_far_from_the_origin(fg, ctx):
         assert_topm_matches(idx_g.cpu().numpy(), resp_g.cpu().numpy(), idx_r, resp_r, next_r, what=f"path {path}, far from the origin")
 
 
+@pytest.mark.parametrize("N,D,K", [(3000, 3, 1), (7001, 3, 5), (2000, 8, 2)])
+def test_forced_tensor_path_small_dimension_far_from_the_origin(fg, ctx, N, D, K):
+    """Few dimensions, few components, data 50 units from the origin: log2 Z of a point is small while the error estimate
+    of the expanded form is not negligible, and the log-likelihood sums that error instead of averaging it out; the limit
+    above which components are recomputed exactly is therefore capped by the dimension."""
+    rng = np.random.default_rng(N + D + K)
+    X = (rng.normal(size=(N, D)) * 0.7 + 50.0).astype(np.float32)
+    mu = (X[rng.integers(0, N, K)] + 0.1 * rng.normal(size=(K, D))).astype(np.float32)
+    var = rng.uniform(0.3, 2.0, size=(K, D)).astype(np.float32)
+    pi = rng.dirichlet(np.ones(K)).astype(np.float32)
+    ref = orc.em_step(X, pi, mu, var)
+    ctx.gmm_set_path(fg.GMM_PATH_TENSOR)
+    for _ in range(2):                      # the second call may run the other filter
+        got = _gpu_step(ctx, _t(X), pi, mu, var)
+        assert abs(got[3] - ref[3]) <= 1e-5 * abs(ref[3])
+        assert_stats_close(N, data_scale(X), got[:3], ref[:3], f"forced tensor path N={N} D={D} K={K}")
+
+
 def test_scratch_does_not_grow_with_n(fg, ctx):
     assert fg.gmm_scratch_bytes(128, 1024) == fg.gmm_scratch_bytes(128, 1024)
     spec = synth.CONFIGS[2]

@@ -1149,7 +1149,7 @@ __global__ void __launch_bounds__(128) tc_prepare_kernel(int D, int K, const flo
                                                          uint32_t* __restrict__ phi_img,
                                                          unsigned char* __restrict__ plo_img, float* __restrict__ tk,
                                                          float* __restrict__ ck, float* __restrict__ illb, float cond_limit,
-                                                         float ll_budget, int* __restrict__ flags, uint32_t* __restrict__ phi_rm,
+                                                         int* __restrict__ flags, uint32_t* __restrict__ phi_rm,
                                                          uint32_t* __restrict__ plo_rm, float2* __restrict__ tkck) {
     const int k = blockIdx.x, d = threadIdx.x;
     const int slice = k >> 7, row = k & 127;
@@ -1218,12 +1218,7 @@ __global__ void __launch_bounds__(128) tc_prepare_kernel(int D, int K, const flo
         // conditioning estimate of the expanded form: 2^-22 sum_d w2 * 3 (mu^2 + 9 var) ~ absolute log2 error bound
         const double cond = red_cond[0] * 2.384185791015625e-07;
         float margin = 0.f;
-        // The log-likelihood does not average a component's error out over its points: it sums it, weighted by the
-        // component's share of the points.  Components are therefore also flagged when cond_k > ll_budget / (pi_k K), which
-        // keeps sum_k pi_k cond_k over the unflagged ones below ll_budget (0: no such rule).
-        double limit_k = (double)cond_limit;
-        if (k < K && ll_budget > 0.f && pi[k] > 0.f) limit_k = fmin(limit_k, (double)ll_budget / ((double)pi[k] * (double)K));
-        if (k < K && cond > limit_k) {
+        if (k < K && cond > (double)cond_limit) {
             margin = (float)fmin(8.0 * cond, 1e30);       // E_k: error bound of the approximate log2 z (8 x the estimate)
             atomicOr(flags, 1);
             atomicAdd(flags + 4, 1);                      // how many: the tile kernel picks its filter by their share
@@ -1422,7 +1417,7 @@ TcPlan tc_plan(int D, int K, int num_sms) {
 }
 
 cudaError_t launch_prepare_tc(cudaStream_t s, int D, int K, const float* pi, const float* mu, const float* var,
-                              const TcBuffers& tb, float cond_limit, float ll_budget, int* status, bool ill_list) {
+                              const TcBuffers& tb, float cond_limit, int* status, bool ill_list) {
     const TcPlan pl = tc_plan(D, K, 148);
     (void)status;
     cudaError_t e0 = cudaMemsetAsync(tb.flags, 0, 8 * sizeof(int), s);
@@ -1430,7 +1425,7 @@ cudaError_t launch_prepare_tc(cudaStream_t s, int D, int K, const float* pi, con
     tc_scale_kernel<<<128, 128, 0, s>>>(D, K, pi, mu, var, tb.sd, tb.kap);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    tc_prepare_kernel<<<pl.Kpad, 128, 0, s>>>(D, K, pi, mu, var, tb.sd, tb.kap, tb.phi_img, tb.plo_img, tb.tk, tb.ck, tb.illb, cond_limit, ll_budget, tb.flags,
+    tc_prepare_kernel<<<pl.Kpad, 128, 0, s>>>(D, K, pi, mu, var, tb.sd, tb.kap, tb.phi_img, tb.plo_img, tb.tk, tb.ck, tb.illb, cond_limit, tb.flags,
                                                   reinterpret_cast<uint32_t*>(tb.p_hi_rm), reinterpret_cast<uint32_t*>(tb.p_lo_rm),
                                                   reinterpret_cast<float2*>(tb.tkck));
     e = cudaGetLastError();

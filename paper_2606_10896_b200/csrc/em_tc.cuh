@@ -66,7 +66,7 @@ void tc_set_test_hooks(int silent_rank, unsigned long long wait_limit_ns);
 TcPlan tc_plan(int D, int K, int num_sms);
 cudaError_t tc_max_clusters(int D, int K, int* out);
 cudaError_t launch_prepare_tc(cudaStream_t s, int D, int K, const float* pi, const float* mu, const float* var,
-                              const TcBuffers& tb, float cond_limit, float ll_budget, int* status, bool ill_list = false);
+                              const TcBuffers& tb, float cond_limit, int* status, bool ill_list = false);
 // One pass over at most TC_YPOINTS points: X -> the two fp16 planes of Y in scratch (read by the tile kernel through TMA).
 cudaError_t launch_transform_tc(cudaStream_t s, const float* X, int64_t n, int D, const TcBuffers& tb);
 // n <= TC_YPOINTS points whose planes launch_transform_tc has written.

@@ -306,8 +306,7 @@ int prepare_and_choose(gmm_ctx* ctx, int64_t N, int D, int K, const float* pi, c
     // about 0.72 D in size, so for small D (where little else is large) the limit is capped at 4e-5 D, which keeps the
     // log-likelihood within 1e-5 relative; at D >= 32 typical estimates (1e-3) are 1e-5 of log2 Z without a cap.
     if (ctx->tc_cond_limit < 0.f && D < 32) limit = std::fmin(limit, 4e-5f * (float)D);
-    const float ll_budget = 0.f;      // (the kernel's pi-weighted rule: off; it flags well-populated components, at great cost)
-    KL(launch_prepare_tc(ctx->stream, D, K, pi, mu, var, ctx->tc(), limit, ll_budget, &ctx->result()->status));
+    KL(launch_prepare_tc(ctx->stream, D, K, pi, mu, var, ctx->tc(), limit, &ctx->result()->status));
     ctx->launches += 2;   // launch_prepare_tc enqueues three kernels
     // the number of ill-conditioned components travels back with the result: the next step picks its filter by it
     CU(cudaMemcpyAsync(&ctx->result()->n_ill, ctx->tc().flags + 4, sizeof(int), cudaMemcpyDeviceToDevice, ctx->stream));
@@ -685,7 +684,7 @@ int assign_topm_impl(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, cons
     if (tensor) {
         const TcBuffers tb = ctx->tc();
         const float limit = ctx->tc_cond_limit >= 0.f ? ctx->tc_cond_limit : 0.01f;
-        KL(launch_prepare_tc(ctx->stream, D, K, pi, mu, var, tb, limit, 0.f, &ctx->result()->status, true));
+        KL(launch_prepare_tc(ctx->stream, D, K, pi, mu, var, tb, limit, &ctx->result()->status, true));
         ctx->launches += 3;
         KL(launch_ill_cache_tc(ctx->stream, D, mu, ctx->w2(), ctx->c2(), tb));
         const int64_t piece = ctx->tc_piece;

@@ -445,10 +445,23 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                     // which every value reaches, also the -inf of a padded component)
                     const bool flagged = illb > 0.f;
                     const float reach = illb + ILL_MARGIN;
+                    // Cheapest first: a value that does not reach the LOWEST of the 32 bounds reaches none (5 shuffles and
+                    // no per-point shuffle; collapsed components, hopeless for all points of most tiles, end here).
+                    float lbmin = lb_own;
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const float lbj = __shfl_sync(0xffffffffu, lb_own, j);
-                        if (flagged && j < nvalid && l[j] + reach >= lbj) mlo |= 1u << j;
+                    for (int o = 16; o > 0; o >>= 1) lbmin = fminf(lbmin, __shfl_xor_sync(0xffffffffu, lbmin, o));
+                    bool maybe = false;
+                    if (flagged) {
+                        const float cut = lbmin - reach;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) maybe |= l[j] >= cut;
+                    }
+                    if (__any_sync(0xffffffffu, maybe)) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const float lbj = __shfl_sync(0xffffffffu, lb_own, j);
+                            if (flagged && j < nvalid && l[j] + reach >= lbj) mlo |= 1u << j;
+                        }
                     }
                     // For a component that is narrow in a few dimensions only, E is in the thousands and almost every pair
                     // passes that test.  Such pairs are then tested exactly: c_k minus the terms of the component's 8

@@ -169,6 +169,27 @@ int gmm_build_posting_lists(gmm_ctx* ctx, const int32_t* idx, const float* resp,
 int gmm_kmeans_step(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const float* centroids,
                     int32_t* assign, int32_t* work, float* centroids_out, int64_t* counts, double* inertia);
 
+/* Fisher-vector encoding of G groups of points under a fixed mixture: the per-group use of the fused pattern (log-sum-exp
+ * over the K weighted Gaussian terms, then responsibility-weighted statistics) that the paper's Discussion (Section 6)
+ * names.  The paper prints no formula; the standard definition is used.  For a group of T points with responsibilities
+ * r_tk (Section 2),
+ *   G_mu[k, d]    = 1 / (T sqrt(pi_k))   * sum_t r_tk (x_td - mu_kd) / sigma_kd
+ *   G_sigma[k, d] = 1 / (T sqrt(2 pi_k)) * sum_t r_tk ((x_td - mu_kd)^2 / sigma_kd^2 - 1),   sigma_kd = sqrt(var_kd),
+ * i.e. the gradient of the group's mean log-likelihood in (mu, sigma), each coordinate divided by the square root of
+ * its diagonal Fisher information.  Each group's (N_k, S1, S2) come from the tile kernels of gmm_em_step (nothing of
+ * size T x K is written to memory) and are turned into the two parts in float64.
+ *   X [N x D]: device, row-major fp32; group g is rows offsets[g] .. offsets[g + 1] - 1.
+ *   offsets [G + 1] int64, HOST: non-decreasing, offsets[0] >= 0, offsets[G] <= N; an empty group gets zeros.
+ *   pi [K], mu [K x D], var [K x D]: device fp32, as for gmm_em_step; a component with pi_k = 0 gets zeros.
+ *   fv [G x 2 x K x D] fp32, device out: per group the means part [K x D], then the standard-deviations part [K x D].
+ *   No power or L2 normalisation is applied.
+ *   loglik (host out, may be NULL): the total log-likelihood of all the groups' points.
+ * Accuracy: that of the statistics (about 1e-6 of the data scale, relative to N_k), so a coordinate is exact to about
+ * 1e-5 (1 + |G|) when |mu| / sigma is moderate; data far from the origin in units of sigma should be centred first.
+ * Errors as gmm_em_step; GMM_EINVAL for offsets out of order or out of range.  Synchronises the stream. */
+int gmm_fisher_vectors(gmm_ctx* ctx, const float* X, int64_t N, const int64_t* offsets, int G, int D, int K,
+                       const float* pi, const float* mu, const float* var, float* fv, double* loglik);
+
 /* The statistics of gmm_em_step for callers that cannot allocate device memory.  (The paper has no counterpart of
  * this entry point; it exists for the library's users.)
  *

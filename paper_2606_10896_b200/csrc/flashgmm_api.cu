@@ -864,6 +864,64 @@ int gmm_kmeans_step(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const
     return GMM_OK;
 }
 
+int gmm_fisher_vectors(gmm_ctx* ctx, const float* X, int64_t N, const int64_t* offsets, int G, int D, int K,
+                       const float* pi, const float* mu, const float* var, float* fv, double* loglik) {
+    CHECK(check_shape(ctx, N, D, K));
+    CHECK(check_ptr(ctx, X, 4, "X"));
+    CHECK(check_ptr(ctx, pi, 4, "pi"));
+    CHECK(check_ptr(ctx, mu, 4, "mu"));
+    CHECK(check_ptr(ctx, var, 4, "var"));
+    CHECK(check_ptr(ctx, fv, 4, "fv"));
+    if (!offsets) return fail(ctx, GMM_EINVAL, "offsets is NULL");
+    if (G < 1) return fail(ctx, GMM_EINVAL, "G must be >= 1 (got %d)", G);
+    int64_t smallest = 0;                       // size of the smallest group that has points
+    for (int g = 0; g < G; ++g) {
+        if (offsets[g] < 0 || offsets[g + 1] < offsets[g] || offsets[g + 1] > N)
+            return fail(ctx, GMM_EINVAL, "offsets[%d..%d] = %lld, %lld: must be non-decreasing inside [0, N]", g, g + 1,
+                        (long long)offsets[g], (long long)offsets[g + 1]);
+        const int64_t T = offsets[g + 1] - offsets[g];
+        if (T > 0 && (smallest == 0 || T < smallest)) smallest = T;
+    }
+    DeviceGuard guard(ctx->device);
+    CHECK(ensure_scratch(ctx, D, K));
+    const size_t KD = (size_t)K * D;
+    double* Nk = ctx->stats();
+    double* S1 = Nk + K;
+    double* S2 = S1 + KD;
+    // One preparation for all groups.  The conditioning limit of the tensor path follows the points per component of the
+    // smallest group: a group's statistics are averaged over its own points only.
+    int path;
+    CHECK(prepare_and_choose(ctx, smallest > 0 ? smallest : 1, D, K, pi, mu, var, &path));
+    CU(cudaMemsetAsync(&ctx->result()->ll[0], 0, 8, ctx->stream));
+    for (int g = 0; g < G; ++g) {
+        const int64_t T = offsets[g + 1] - offsets[g];
+        float* out = fv + (size_t)g * 2 * KD;
+        if (T == 0) {
+            CU(cudaMemsetAsync(out, 0, 2 * KD * sizeof(float), ctx->stream));
+            continue;
+        }
+        CU(cudaMemsetAsync(Nk, 0, ((size_t)K + 2 * KD) * 8, ctx->stream));
+        CHECK(accumulate_points(ctx, path, X + offsets[g] * D, T, D, K, mu, Nk, S1, S2, 0));
+        KL(launch_fisher(ctx->stream, T, D, K, Nk, S1, S2, pi, mu, var, out));
+    }
+    ctx->last_path = path;
+    double total = 0.0;
+    if (smallest == 0) {                        // no points at all: nothing was accumulated, only the parameters were checked
+        DevResult r;
+        CU(cudaMemcpyAsync(&r, ctx->result(), sizeof(DevResult), cudaMemcpyDeviceToHost, ctx->stream));
+        CU(cudaStreamSynchronize(ctx->stream));
+        if (r.status & ST_BAD_VAR) return fail(ctx, GMM_ENUMERIC, "var must be finite and > 0");
+        if (r.status & ST_BAD_PI) return fail(ctx, GMM_ENUMERIC, "pi must be finite and >= 0");
+        if (r.status & ST_NONFINITE) return fail(ctx, GMM_ENUMERIC, "non-finite parameter");
+        if (loglik) *loglik = 0.0;
+        return GMM_OK;
+    }
+    const int rc = read_result(ctx, 0, &total);
+    if (rc != GMM_OK) return rc;
+    if (loglik) *loglik = total;
+    return GMM_OK;
+}
+
 const char* gmm_strerror(int code) {
     switch (code) {
         case GMM_OK: return "ok";

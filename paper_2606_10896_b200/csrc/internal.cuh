@@ -60,6 +60,11 @@ cudaError_t launch_finalize(cudaStream_t s, int64_t N, int D, int K, const doubl
 cudaError_t launch_finalize_isotropic(cudaStream_t s, int64_t N, int D, int K, const double* Nk, const double* S1,
                                       const double* S2, float var_floor, float* pi, float* mu, float* var);
 
+// ---- Fisher vector of one group from its statistics (paper Section 6) ----------------------------------------------
+// out[2 * K * D] (device): the means part [K x D], then the standard-deviations part [K x D]
+cudaError_t launch_fisher(cudaStream_t s, int64_t T, int D, int K, const double* Nk, const double* S1, const double* S2,
+                          const float* pi, const float* mu, const float* var, float* out);
+
 // ---- IVF posting lists from the top-m assignment (paper Sections 4.2-4.3) ---------------------------------------
 constexpr int PL_MAX_BLOCKS = 1024;       // the vectors are cut into at most this many contiguous ranges
 constexpr int PL_MAX_K = 8192;            // one 32-bit cursor per cluster in shared memory

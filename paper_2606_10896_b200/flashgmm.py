@@ -57,6 +57,9 @@ EXPORTS = {
     "gmm_kmeans_step": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_int, ctypes.c_void_p,
                                        ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                        ctypes.POINTER(ctypes.c_double)]),
+    "gmm_fisher_vectors": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p, ctypes.c_int,
+                                          ctypes.c_int, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                          ctypes.c_void_p, ctypes.POINTER(ctypes.c_double)]),
     "gmm_em_step_static": (ctypes.c_int, [ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int,
                                           ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                           ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
@@ -304,6 +307,24 @@ class Context:
                                          ctypes.byref(total), ctypes.byref(mean))
         self._check(rc)
         return offsets, items, int(total.value), float(mean.value)
+
+    def gmm_fisher_vectors(self, X, offsets, pi, mu, var, out=None):
+        """Fisher vectors of the groups of consecutive rows given by ``offsets`` (host int64 [G + 1]):
+        (fv float32 [G, 2, K, D], total log-likelihood)."""
+        N, D = X.shape
+        K = mu.shape[0]
+        offsets = np.ascontiguousarray(offsets, dtype=np.int64)
+        if offsets.ndim != 1 or offsets.shape[0] < 2:
+            raise ValueError("offsets must hold G + 1 >= 2 entries")
+        G = offsets.shape[0] - 1
+        fv = out if out is not None else torch.empty((G, 2, K, D), dtype=torch.float32, device=X.device)
+        ll = ctypes.c_double(0.0)
+        rc = lib.gmm_fisher_vectors(self._h, _dev(X, torch.float32, (N, D), "X"), N, _host(offsets, np.int64, (G + 1,), "offsets"),
+                                    G, D, K, _dev(pi, torch.float32, (K,), "pi"), _dev(mu, torch.float32, (K, D), "mu"),
+                                    _dev(var, torch.float32, (K, D), "var"), _dev(fv, torch.float32, (G, 2, K, D), "fv"),
+                                    ctypes.byref(ll))
+        self._check(rc)
+        return fv, float(ll.value)
 
     def gmm_kmeans_step(self, X, centroids, out=None, work=None):
         """One Lloyd iteration: (assign int32 [N], new centroids float32 [K, D], counts int64 [K], inertia)."""

@@ -240,6 +240,10 @@ struct TcKernelParams {
     XSlot* xg;                     // [Q][4][CL][64] exchange slots (zeroed before every launch)
     XSlot* xl;                     // [Q][4][CL][4][64] lower-bound slots, one per warp and point
     int* status;
+    // Grouped launches (one group of points per CTA group, e.g. Fisher vectors): tile t of the planes holds tile_valid[t]
+    // points (0 .. BN; the rest of its rows are zeros) taken from rows tile_src[t] .. of X.  Both NULL otherwise.
+    const int* tile_valid;
+    const int64_t* tile_src;
 #ifdef FLASHGMM_DEBUG
     float* dbg;      // [Kpad][64] log2 z of the first tile
     int dbg_cluster, dbg_i; // which (group, local tile) the logit dump records
@@ -367,7 +371,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
             const uint32_t ph = (uint32_t)((i >> 1) & 1);
             const int64_t tile = cluster_id + i * p.Q;
             const int64_t row0 = tile * BN;
-            const int nvalid = (int)((p.n - row0 < BN) ? (p.n - row0) : BN) - p0;     // valid points of this group's half
+            const int tile_points = p.tile_valid ? __ldg(p.tile_valid + tile) : (int)((p.n - row0 < BN) ? (p.n - row0) : BN);
+            const int nvalid = tile_points - p0;                                      // valid points of this group's half
+            const int64_t xrow0 = p.tile_src ? __ldg(p.tile_src + tile) : row0;       // where the tile's points sit in X
 
             TIC(tk_);
             if (!bar_wait(BAR(B_LFULL0 + s), ph, abort_flag, p.status, false)) alive = false;
@@ -584,7 +590,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
 #ifdef FLASHGMM_DEBUG
                         if (p.dbg_clk && blockIdx.x == 0 && lane == 0) atomicAdd((unsigned long long*)&p.dbg_clk[25], 1ull);
 #endif
-                        const float* xr = p.X + (row0 + p0 + j) * p.D;
+                        const float* xr = p.X + (xrow0 + p0 + j) * p.D;
                         const float* mr = p.mu + (size_t)kk * p.D;
                         const float* wr = p.w2 + (size_t)kk * p.D;
                         float q = 0.f;
@@ -1062,7 +1068,7 @@ __device__ __forceinline__ void tc_load_unit(const float* __restrict__ X, int64_
     }
 }
 
-__device__ __forceinline__ void tc_store_unit(const float (&x)[8], int64_t n, const float* __restrict__ sd,
+__device__ __forceinline__ void tc_store_unit(const float (&x)[8], bool valid, const float* __restrict__ sd,
                                               const float* __restrict__ kap, int64_t u, unsigned char* __restrict__ yhi,
                                               unsigned char* __restrict__ ylo) {
     const int64_t row = u >> 4;
@@ -1074,7 +1080,7 @@ __device__ __forceinline__ void tc_store_unit(const float (&x)[8], int64_t n, co
         u0 = fminf(fmaxf(u0, -240.f), 240.f);
         u1 = fminf(fmaxf(u1, -240.f), 240.f);
         float q0 = fmaf(u0, u0, __ldg(kap + d0 + j)), q1 = fmaf(u1, u1, __ldg(kap + d0 + j + 1));
-        if (row >= n) { q0 = 0.f; q1 = 0.f; }
+        if (!valid) { q0 = 0.f; q1 = 0.f; }
         const __half2 h = __floats2half2_rn(u0, u1);
         const float2 hf = __half22float2(h);
         const __half2 g2 = __floats2half2_rn(u0 - hf.x, u1 - hf.y);
@@ -1105,8 +1111,31 @@ __global__ void __launch_bounds__(256) tc_transform_kernel(const float* __restri
         float xa[8], xb[8];
         tc_load_unit(X, n, D, vec_ok, u, units, xa);
         tc_load_unit(X, n, D, vec_ok, u + stride, units, xb);
-        tc_store_unit(xa, n, sd, kap, u, yhi, ylo);
-        if (u + stride < units) tc_store_unit(xb, n, sd, kap, u + stride, yhi, ylo);
+        tc_store_unit(xa, (u >> 4) < n, sd, kap, u, yhi, ylo);
+        if (u + stride < units) tc_store_unit(xb, ((u + stride) >> 4) < n, sd, kap, u + stride, yhi, ylo);
+    }
+}
+
+// The same planes for a grouped launch: row r of the planes belongs to tile t = r / BN and holds point
+// tile_src[t] + (r mod BN) of X if (r mod BN) < tile_valid[t], zeros otherwise.
+__global__ void __launch_bounds__(256) tc_transform_grouped_kernel(const float* __restrict__ X, int64_t rows, int D,
+                                                                   const int* __restrict__ tile_valid,
+                                                                   const int64_t* __restrict__ tile_src,
+                                                                   const float* __restrict__ sd, const float* __restrict__ kap,
+                                                                   unsigned char* __restrict__ yhi, unsigned char* __restrict__ ylo) {
+    const int64_t units = rows * 16;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; u < units; u += stride) {
+        const int64_t row = u >> 4;
+        const int64_t t = row / BN;
+        const int j = (int)(row - t * BN);
+        const bool valid = j < __ldg(tile_valid + t);
+        const float* xr = X + (valid ? (__ldg(tile_src + t) + j) * D : 0);
+        const int d0 = (int)(u & 15) * 8;
+        float x[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) x[q] = (valid && d0 + q < D) ? __ldg(xr + d0 + q) : 0.f;
+        tc_store_unit(x, valid, sd, kap, u, yhi, ylo);
     }
 }
 
@@ -1390,7 +1419,58 @@ __global__ void tc_reduce_kernel(int D, int K, int Kpad, int Q, const double* __
     *dst = accumulate ? (*dst + s) : s;
 }
 
+// Fisher vectors of the groups of a grouped launch, straight from the per-CTA-group partials (group b of the launch =
+// CTA group b): the statistics are unscaled as in tc_reduce_kernel, then
+//   G_mu = (S1 - mu N_k) / (T sigma sqrt(pi)),  G_sigma = (S2 - 2 mu S1 + (mu^2 - var) N_k) / (T var sqrt(2 pi))
+// in float64.  out_index[b] = which of the caller's groups it is, group_points[b] = its T.
+__global__ void tc_fisher_kernel(int D, int K, int Kpad, const double* __restrict__ partial, const float* __restrict__ sd,
+                                 const float* __restrict__ kap, const float* __restrict__ pi, const float* __restrict__ mu,
+                                 const float* __restrict__ var, const int* __restrict__ out_index,
+                                 const int64_t* __restrict__ group_points, float* __restrict__ fv) {
+    const size_t KD = (size_t)K * D;
+    const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= KD) return;
+    const int b = blockIdx.y;
+    const int k = (int)(e / D), d = (int)(e % D);
+    const double* pb = partial + (size_t)b * TC_PCOLS * Kpad;
+    const int col = 16 * (d >> 3) + (d & 7);
+    const double unscale = 1.0 / (double)TC_RSCALE;
+    const double s = (double)sd[d];
+    const double nk_raw = pb[(size_t)256 * Kpad + k] + pb[(size_t)257 * Kpad + k];
+    const double nk = nk_raw * unscale;
+    const double s1 = pb[(size_t)col * Kpad + k] * unscale / s;
+    const double s2 = (pb[(size_t)(col + 8) * Kpad + k] - (double)kap[d] * nk_raw) * unscale / (s * s);
+    const double w = (double)pi[k], t = (double)group_points[b];
+    float gm = 0.f, gs = 0.f;
+    if (w > 0.0) {
+        const double m = (double)mu[e], v = (double)var[e];
+        gm = (float)((s1 - m * nk) / (t * sqrt(v) * sqrt(w)));
+        gs = (float)(((s2 - 2.0 * m * s1) + (m * m - v) * nk) / (t * v * sqrt(2.0 * w)));
+    }
+    float* out = fv + (size_t)out_index[b] * 2 * KD;
+    out[e] = gm;
+    out[KD + e] = gs;
+}
+
 }  // namespace
+
+cudaError_t launch_fisher_tc(cudaStream_t s, int D, int K, int groups, const TcBuffers& tb, const float* pi, const float* mu,
+                             const float* var, const int* out_index, const int64_t* group_points, float* fv) {
+    const TcPlan pl = tc_plan(D, K, 148);
+    const size_t n = (size_t)K * D;
+    tc_fisher_kernel<<<dim3((unsigned)((n + 255) / 256), (unsigned)groups), 256, 0, s>>>(D, K, pl.Kpad, tb.partial, tb.sd, tb.kap, pi, mu,
+                                                                                       var, out_index, group_points, fv);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_transform_grouped_tc(cudaStream_t s, const float* X, int64_t rows, int D, const int* tile_valid,
+                                        const int64_t* tile_src, const TcBuffers& tb) {
+    if (rows < 1 || rows > TC_YPOINTS || rows % TC_BN != 0) return cudaErrorInvalidValue;
+    int64_t blocks = (rows * 16 + 255) / 256;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    tc_transform_grouped_kernel<<<(unsigned)blocks, 256, 0, s>>>(X, rows, D, tile_valid, tile_src, tb.sd, tb.kap, tb.y_hi, tb.y_lo);
+    return cudaGetLastError();
+}
 
 #ifdef FLASHGMM_DEBUG
 float* g_tc_debug = nullptr;
@@ -1502,10 +1582,12 @@ cudaError_t set_smem_attr(bool big, bool tight) {
 }  // namespace
 
 cudaError_t launch_em_tc(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu, const float* w2,
-                         const float* c2, const TcBuffers& tb, int Q, int flush_tiles, bool tight, int* status) {
+                         const float* c2, const TcBuffers& tb, int Q, int flush_tiles, bool tight, int* status,
+                         const int* tile_valid, const int64_t* tile_src) {
     const TcPlan pl = tc_plan(D, K, 148);
     const bool big = pl.CL > 8;
     TcKernelParams p;
+    p.tile_valid = tile_valid; p.tile_src = tile_src;
     p.X = X; p.n = n; p.D = D; p.K = K; p.CL = pl.CL; p.Q = Q; p.n_ks = pl.n_ks;
     p.flush = (flush_tiles < 2) ? 2 : (flush_tiles & ~1);
     p.order = g_tc_order;

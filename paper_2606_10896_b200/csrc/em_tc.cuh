@@ -73,7 +73,17 @@ cudaError_t launch_transform_tc(cudaStream_t s, const float* X, int64_t n, int D
 // mu, w2, c2: the FP32 path's derived parameters (launch_prepare_fp32), used to recompute ill-conditioned logits exactly.
 // tight: use the filter meant for launches in which many components are ill-conditioned (tb.flags[4] counts them).
 cudaError_t launch_em_tc(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu, const float* w2,
-                         const float* c2, const TcBuffers& tb, int Q, int flush_tiles, bool tight, int* status);
+                         const float* c2, const TcBuffers& tb, int Q, int flush_tiles, bool tight, int* status,
+                         const int* tile_valid = nullptr, const int64_t* tile_src = nullptr);
+// Grouped launches: CTA group b of a launch with Q = `groups` takes the tiles b, b + Q, b + 2 Q, ... of the planes, so a
+// plane layout in which those tiles hold the points of one group of the caller (an image's descriptors, say) leaves that
+// group's statistics in partial[b].  tile_valid[t] (0 .. TC_BN) = points of tile t, tile_src[t] = their first row in X
+// (device arrays, rows / TC_BN entries); launch_em_tc then gets n = rows and the same two arrays.
+cudaError_t launch_transform_grouped_tc(cudaStream_t s, const float* X, int64_t rows, int D, const int* tile_valid,
+                                        const int64_t* tile_src, const TcBuffers& tb);
+// After a grouped launch_em_tc: Fisher vector of group b (its T = group_points[b]) into fv[out_index[b]][2][K][D].
+cudaError_t launch_fisher_tc(cudaStream_t s, int D, int K, int groups, const TcBuffers& tb, const float* pi, const float* mu,
+                             const float* var, const int* out_index, const int64_t* group_points, float* fv);
 // After launch_prepare_tc(..., ill_list = true): fills tb.ill_cache for the first min(flags[2], TC_MAX_ILL) listed components.
 // w2, c2: the FP32 path's derived parameters (launch_prepare_fp32).
 cudaError_t launch_ill_cache_tc(cudaStream_t s, int D, const float* mu, const float* w2, const float* c2, const TcBuffers& tb);

@@ -3,6 +3,7 @@
 #include "internal.cuh"
 #include "em_tc.cuh"
 
+#include <algorithm>
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
@@ -100,6 +101,8 @@ struct gmm_ctx {
     void* km_scratch = nullptr;      // k-means step: list offsets, per-segment float64 sums
     void* at_scratch = nullptr;      // tensor-core assignment: candidate records of one piece of points
     size_t at_scratch_bytes = 0;
+    void* fv_scratch = nullptr;      // Fisher vectors, grouped launches: tile and group tables
+    size_t fv_scratch_bytes = 0;
     void* km_unit = nullptr;         // k-means step on the tensor path: var = 1 [K x D], pi = 1 / K [K]
     size_t km_unit_bytes = 0;
     size_t km_scratch_bytes = 0;
@@ -444,6 +447,7 @@ int gmm_destroy(gmm_ctx* ctx) {
     if (ctx->pl_scratch) cudaFree(ctx->pl_scratch);
     if (ctx->km_scratch) cudaFree(ctx->km_scratch);
     if (ctx->at_scratch) cudaFree(ctx->at_scratch);
+    if (ctx->fv_scratch) cudaFree(ctx->fv_scratch);
     if (ctx->km_unit) cudaFree(ctx->km_unit);
     if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
     if (ctx->ev_created)
@@ -888,12 +892,105 @@ int gmm_fisher_vectors(gmm_ctx* ctx, const float* X, int64_t N, const int64_t* o
     double* Nk = ctx->stats();
     double* S1 = Nk + K;
     double* S2 = S1 + KD;
-    // One preparation for all groups.  The conditioning limit of the tensor path follows the points per component of the
-    // smallest group: a group's statistics are averaged over its own points only.
+    // One preparation for all groups.  The conditioning limit of the tensor path is the one an EM step over all the
+    // groups' points would use: what bounds the accuracy of a Fisher coordinate is the cancellation between the raw
+    // moments (N_k, S1, S2), about 4e-6 (1 + mu^2 / var) N_k / (T sqrt(pi_k)), which the stricter limit of the smallest
+    // group alone would not improve (measured: the same errors with and without any exact recomputation).
     int path;
-    CHECK(prepare_and_choose(ctx, smallest > 0 ? smallest : 1, D, K, pi, mu, var, &path));
+    int64_t total_points = 0;
+    for (int g = 0; g < G; ++g) total_points += offsets[g + 1] - offsets[g];
+    CHECK(prepare_and_choose(ctx, total_points > 0 ? total_points : 1, D, K, pi, mu, var, &path));
+    if (path == GMM_PATH_TENSOR && ctx->path == GMM_PATH_AUTO) {
+        // Once the limit flags nearly all the components the tile kernel has no well-conditioned logits left to bound
+        // a point's maximum with, tests every pair exactly, and the FP32 kernels are the faster exact path.
+        int n_ill = 0;
+        CU(cudaMemcpyAsync(&n_ill, ctx->tc().flags + 4, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
+        CU(cudaStreamSynchronize(ctx->stream));
+        ctx->tc_n_ill = n_ill;
+        if ((int64_t)n_ill * 50 > (int64_t)K * 49) path = GMM_PATH_FP32;
+    }
     CU(cudaMemsetAsync(&ctx->result()->ll[0], 0, 8, ctx->stream));
+    // Tensor path: groups small enough that one launch can hold a tile column for each of its CTA groups are processed
+    // several at a time, CTA group b of a launch accumulating the statistics of one of them (its tiles are laid out at
+    // b, b + Q, ... in the planes); their vectors come straight from the per-CTA-group partials.  Groups are taken in
+    // order of size so that the groups of a launch finish together.  Larger groups go one at a time through the step's
+    // own accumulation below.
+    std::vector<char> batched((size_t)G, 0);
+    if (path == GMM_PATH_TENSOR) {
+        const TcBuffers tb = ctx->tc();
+        const TcPlan pl = tc_plan(D, K, 160);
+        const int Qmax = ctx->tc_Q;
+        const int64_t cap_tiles = ctx->tc_piece / TC_BN;                        // tiles that the planes of one launch hold
+        std::vector<int> order;
+        for (int g = 0; g < G; ++g) {
+            const int64_t T = offsets[g + 1] - offsets[g];
+            if (T > 0 && 2 * ((T + TC_BN - 1) / TC_BN) <= cap_tiles) order.push_back(g);      // at least two per launch
+        }
+        std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
+            return offsets[a + 1] - offsets[a] > offsets[b + 1] - offsets[b];
+        });
+        struct Batch { size_t tile0, group0; int Q; int64_t tiles_each; };
+        std::vector<Batch> batches;
+        std::vector<int> h_valid, h_index;
+        std::vector<int64_t> h_src, h_points;
+        for (size_t a = 0; a < order.size();) {
+            const int64_t T0 = offsets[order[a] + 1] - offsets[order[a]];          // the largest of the batch
+            const int64_t tiles_each = (T0 + TC_BN - 1) / TC_BN;
+            const int Qb = (int)std::min<int64_t>(std::min<int64_t>(Qmax, cap_tiles / tiles_each), (int64_t)(order.size() - a));
+            // A launch of Qb < Qmax groups leaves CTA groups idle; a group on its own uses them all but pays about 30
+            // tile times of launches and reductions.  Per group: tiles / Qb against tiles / Qmax + 30.
+            if (Qb < 2 || tiles_each * (Qmax - Qb) > (int64_t)30 * Qb * Qmax) { ++a; continue; }      // left to the loop over single groups
+            batches.push_back({h_valid.size(), h_index.size(), Qb, tiles_each});
+            for (int64_t i = 0; i < tiles_each; ++i)
+                for (int b = 0; b < Qb; ++b) {                                     // tile b + i Qb of the planes
+                    const int g = order[a + b];
+                    const int64_t T = offsets[g + 1] - offsets[g];
+                    const int64_t left = T - i * TC_BN;
+                    h_valid.push_back(left <= 0 ? 0 : (int)std::min<int64_t>(left, TC_BN));
+                    h_src.push_back(left <= 0 ? offsets[g] : offsets[g] + i * TC_BN);
+                }
+            for (int b = 0; b < Qb; ++b) {
+                const int g = order[a + b];
+                h_index.push_back(g);
+                h_points.push_back(offsets[g + 1] - offsets[g]);
+                batched[g] = 1;
+            }
+            a += (size_t)Qb;
+        }
+        if (!batches.empty()) {
+            const size_t nt = h_valid.size(), ng = h_index.size();
+            const size_t o_src = 0, o_points = o_src + align256(nt * 8), o_valid = o_points + align256(ng * 8),
+                         o_index = o_valid + align256(nt * 4), total_bytes = o_index + align256(ng * 4);
+            CHECK(grow_buffer(ctx, &ctx->fv_scratch, &ctx->fv_scratch_bytes, total_bytes, "the tile tables of the grouped launches"));
+            unsigned char* base = static_cast<unsigned char*>(ctx->fv_scratch);
+            // (pageable sources: each copy has left the host array when the call returns)
+            CU(cudaMemcpyAsync(base + o_src, h_src.data(), nt * 8, cudaMemcpyHostToDevice, ctx->stream));
+            CU(cudaMemcpyAsync(base + o_points, h_points.data(), ng * 8, cudaMemcpyHostToDevice, ctx->stream));
+            CU(cudaMemcpyAsync(base + o_valid, h_valid.data(), nt * 4, cudaMemcpyHostToDevice, ctx->stream));
+            CU(cudaMemcpyAsync(base + o_index, h_index.data(), ng * 4, cudaMemcpyHostToDevice, ctx->stream));
+            const int64_t* d_src = reinterpret_cast<const int64_t*>(base + o_src);
+            const int64_t* d_points = reinterpret_cast<const int64_t*>(base + o_points);
+            const int* d_valid = reinterpret_cast<const int*>(base + o_valid);
+            const int* d_index = reinterpret_cast<const int*>(base + o_index);
+            bool tight = ctx->tc_n_ill > 0 && (smallest < (int64_t)512 * K || (int64_t)ctx->tc_n_ill * 8 > K);
+            if (ctx->tc_force_filter >= 0) tight = ctx->tc_force_filter == 1;
+            for (const Batch& bt : batches) {
+                const int64_t rows = bt.tiles_each * bt.Q * TC_BN;
+                CU(cudaMemsetAsync(tb.partial, 0, (size_t)bt.Q * pl.Kpad * TC_PCOLS * 8, ctx->stream));
+                CU(cudaMemsetAsync(tb.llpart, 0, (size_t)bt.Q * 16, ctx->stream));
+                CHECK(prof_begin(ctx));
+                KL(launch_transform_grouped_tc(ctx->stream, X, rows, D, d_valid + bt.tile0, d_src + bt.tile0, tb));
+                KL(launch_em_tc(ctx->stream, X, rows, D, K, mu, ctx->w2(), ctx->c2(), tb, bt.Q, ctx->tc_flush, tight,
+                                &ctx->result()->status, d_valid + bt.tile0, d_src + bt.tile0));
+                CHECK(prof_end(ctx));
+                KL(launch_reduce_ll(ctx->stream, tb.llpart, 2 * bt.Q, &ctx->result()->ll[0], true));
+                KL(launch_fisher_tc(ctx->stream, D, K, bt.Q, tb, pi, mu, var, d_index + bt.group0, d_points + bt.group0, fv));
+                ctx->launches += 2;
+            }
+        }
+    }
     for (int g = 0; g < G; ++g) {
+        if (batched[g]) continue;
         const int64_t T = offsets[g + 1] - offsets[g];
         float* out = fv + (size_t)g * 2 * KD;
         if (T == 0) {

@@ -41,6 +41,9 @@ def parse():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--path", default="auto", choices=["auto", "fp32", "tensor"])
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--fisher-points", type=int, default=0,
+                    help="also time gmm_fisher_vectors over the first (at most 2M) points of X in groups of this many "
+                         "consecutive points (outside the timed region; reported as 'fisher_vectors'); 0 skips it")
     ap.add_argument("--assign-m", type=int, default=4,
                     help="also time gmm_assign_topm with this m on the same X (after the timed EM steps, outside their "
                          "timed region; reported as 'assign_topm'); 0 skips it")
@@ -292,6 +295,30 @@ def main():
                   "mean_top1_resp": float(resp[:, 0].mean().item())}
         del idx, resp
 
+    # ---- optional: Fisher vectors of groups of consecutive points of the same X, under the same parameters ----
+    fisher = None
+    if args.fisher_points > 0:
+        T = args.fisher_points
+        n_fv = int(min(N, 2_000_000)) // T * T
+        if n_fv >= T:
+            G = n_fv // T
+            offsets = np.arange(G + 1, dtype=np.int64) * T
+            fv = torch.empty((G, 2, K, D), dtype=torch.float32, device=dev)
+            ctx.gmm_fisher_vectors(X, offsets, pi, mu, var, out=fv)       # warm-up (allocates the tile tables)
+            torch.cuda.synchronize()
+            f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            reps = max(1, min(args.steps, 3))
+            f0.record()
+            for _ in range(reps):
+                ctx.gmm_fisher_vectors(X, offsets, pi, mu, var, out=fv)
+            f1.record()
+            torch.cuda.synchronize()
+            f_ms = f0.elapsed_time(f1) / reps
+            fisher = {"groups": G, "points_per_group": T, "ms": f_ms, "points_per_s": n_fv / (f_ms * 1e-3),
+                      "algorithmic_tflops": 8.0 * n_fv * K * D / (f_ms * 1e-3) / 1e12,
+                      "path": "tensor" if ctx.gmm_last_path() == fg.GMM_PATH_TENSOR else "fp32"}
+            del fv
+
     # ---- end to end through the C ABI with HOST buffers (copies inside the timed region) ----
     e2e = None
     if not args.no_e2e:
@@ -363,7 +390,7 @@ def main():
             "point_component_dim_per_s": N_global * K * D / (ms_step * 1e-3),
             "algorithmic_tflops": 8.0 * N_global * K * D / (ms_step * 1e-3) / 1e12,
             "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": int(launches),
-            "clocks": clocks, "scratch_bytes": int(mem_extra), "assign_topm": assign,
+            "clocks": clocks, "scratch_bytes": int(mem_extra), "assign_topm": assign, "fisher_vectors": fisher,
             "loglik_first_last": [trace[0], trace[-1]],
             "paper_context": {"A100_ms_per_iter_N1M": 3755.0 / 30, "A100_ms_per_iter_N100M": 74270.0 / 30},
         }

@@ -1423,33 +1423,57 @@ __global__ void tc_reduce_kernel(int D, int K, int Kpad, int Q, const double* __
 // CTA group b): the statistics are unscaled as in tc_reduce_kernel, then
 //   G_mu = (S1 - mu N_k) / (T sigma sqrt(pi)),  G_sigma = (S2 - 2 mu S1 + (mu^2 - var) N_k) / (T var sqrt(2 pi))
 // in float64.  out_index[b] = which of the caller's groups it is, group_points[b] = its T.
-__global__ void tc_fisher_kernel(int D, int K, int Kpad, const double* __restrict__ partial, const float* __restrict__ sd,
-                                 const float* __restrict__ kap, const float* __restrict__ pi, const float* __restrict__ mu,
-                                 const float* __restrict__ var, const int* __restrict__ out_index,
-                                 const int64_t* __restrict__ group_points, float* __restrict__ fv) {
-    const size_t KD = (size_t)K * D;
-    const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (e >= KD) return;
-    const int b = blockIdx.y;
-    const int k = (int)(e / D), d = (int)(e % D);
+__global__ void __launch_bounds__(256) tc_fisher_kernel(int D, int K, int Kpad, const double* __restrict__ partial,
+                                                        const float* __restrict__ sd, const float* __restrict__ kap,
+                                                        const float* __restrict__ pi, const float* __restrict__ mu,
+                                                        const float* __restrict__ var, const int* __restrict__ out_index,
+                                                        const int64_t* __restrict__ group_points, float* __restrict__ fv) {
+    // A block takes 32 components x 32 dimensions of one group.  The partials are [column][component] (component
+    // fastest), the output is [component][dimension]: the 64 columns of the 32 dimensions (x and x^2 parts) and the two
+    // N_k columns pass through shared memory, so that both the reads and the writes are contiguous per warp.
+    __shared__ double tile[64][33];
+    __shared__ double nk_s[32];
+    const int k0 = blockIdx.x * 32, d0 = blockIdx.y * 32, b = blockIdx.z;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const double* pb = partial + (size_t)b * TC_PCOLS * Kpad;
-    const int col = 16 * (d >> 3) + (d & 7);
-    const double unscale = 1.0 / (double)TC_RSCALE;
-    const double s = (double)sd[d];
-    const double nk_raw = pb[(size_t)256 * Kpad + k] + pb[(size_t)257 * Kpad + k];
-    const double nk = nk_raw * unscale;
-    const double s1 = pb[(size_t)col * Kpad + k] * unscale / s;
-    const double s2 = (pb[(size_t)(col + 8) * Kpad + k] - (double)kap[d] * nk_raw) * unscale / (s * s);
-    const double w = (double)pi[k], t = (double)group_points[b];
-    float gm = 0.f, gs = 0.f;
-    if (w > 0.0) {
-        const double m = (double)mu[e], v = (double)var[e];
-        gm = (float)((s1 - m * nk) / (t * sqrt(v) * sqrt(w)));
-        gs = (float)(((s2 - 2.0 * m * s1) + (m * m - v) * nk) / (t * v * sqrt(2.0 * w)));
+    const bool kin = k0 + lane < Kpad;
+    for (int c = warp; c < 64; c += 8) {
+        const int d = d0 + (c & 31);                                   // c < 32: the x part, else the x^2 part
+        const int col = 16 * (d >> 3) + (d & 7) + ((c >> 5) << 3);
+        tile[c][lane] = (kin && d < 128) ? pb[(size_t)col * Kpad + k0 + lane] : 0.0;
     }
+    if (warp == 0) nk_s[lane] = kin ? pb[(size_t)256 * Kpad + k0 + lane] + pb[(size_t)257 * Kpad + k0 + lane] : 0.0;
+    __syncthreads();
+    const int d = d0 + lane;
+    if (d >= D) return;
+    const size_t KD = (size_t)K * D;
+    // The differences cancel and are formed in float64; the positive scale factors (1 / (T sigma sqrt(pi)) and
+    // 1 / (T var sqrt(2 pi))) are formed in fp32, whose 1e-7 relative error goes straight into the result (float64
+    // divisions and square roots per element would make this kernel arithmetic-bound).
+    const double unscale = 1.0 / (double)TC_RSCALE;
+    const double u1 = unscale / (double)sd[d], u2 = u1 / (double)sd[d], kp = (double)kap[d];
+    const float inv_t = 1.0f / (float)group_points[b];
     float* out = fv + (size_t)out_index[b] * 2 * KD;
-    out[e] = gm;
-    out[KD + e] = gs;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const int kk = warp + 8 * j, k = k0 + kk;
+        if (k >= K) continue;
+        const double nk_raw = nk_s[kk];
+        const double nk = nk_raw * unscale;
+        const double s1 = tile[lane][kk] * u1;
+        const double s2 = (tile[32 + lane][kk] - kp * nk_raw) * u2;
+        const size_t e = (size_t)k * D + d;
+        const float w = pi[k];
+        float gm = 0.f, gs = 0.f;
+        if (w > 0.f) {
+            const float vf = var[e];
+            const double m = (double)mu[e], v = (double)vf;
+            gm = (float)(s1 - m * nk) * (inv_t * rsqrtf(vf) * rsqrtf(w));
+            gs = (float)((s2 - 2.0 * m * s1) + (m * m - v) * nk) * (inv_t * rsqrtf(2.0f * w) / vf);
+        }
+        out[e] = gm;
+        out[KD + e] = gs;
+    }
 }
 
 }  // namespace
@@ -1457,9 +1481,8 @@ __global__ void tc_fisher_kernel(int D, int K, int Kpad, const double* __restric
 cudaError_t launch_fisher_tc(cudaStream_t s, int D, int K, int groups, const TcBuffers& tb, const float* pi, const float* mu,
                              const float* var, const int* out_index, const int64_t* group_points, float* fv) {
     const TcPlan pl = tc_plan(D, K, 148);
-    const size_t n = (size_t)K * D;
-    tc_fisher_kernel<<<dim3((unsigned)((n + 255) / 256), (unsigned)groups), 256, 0, s>>>(D, K, pl.Kpad, tb.partial, tb.sd, tb.kap, pi, mu,
-                                                                                       var, out_index, group_points, fv);
+    tc_fisher_kernel<<<dim3((unsigned)((K + 31) / 32), (unsigned)((D + 31) / 32), (unsigned)groups), 256, 0, s>>>(
+        D, K, pl.Kpad, tb.partial, tb.sd, tb.kap, pi, mu, var, out_index, group_points, fv);
     return cudaGetLastError();
 }
 

@@ -268,3 +268,21 @@ def test_gpu_fisher_vectors_of_a_group_that_sits_on_one_light_component(K, D, T)
     offsets = np.array([0, T, 2 * T, 2 * T + T // 2], np.int64)
     for path in (fg.GMM_PATH_TENSOR, fg.GMM_PATH_FP32):
         _check_against_oracle(X, offsets, pi, mu, var, path)
+
+
+@pytest.mark.gpu
+def test_gpu_fisher_vectors_many_small_groups_beside_a_large_one():
+    # one call that mixes both routes of the tensor path: 60 groups of 0 .. 3000 points share launches (several groups
+    # per launch, sorted by size), the group of 60,000 points is accumulated on its own
+    from paper_2606_10896_b200 import flashgmm as fg
+
+    rng = np.random.Generator(np.random.PCG64(2024))
+    sizes = [int(v) for v in rng.integers(1, 3000, 60)]
+    sizes[7] = 0
+    sizes[20] = 60000
+    sizes[41] = 64
+    sizes[42] = 65
+    X, offsets, pi, mu, var = _gpu_case(5, 128, 32, sizes)
+    G, used = _check_against_oracle(X, offsets, pi, mu, var)
+    assert used == fg.GMM_PATH_TENSOR
+    assert np.all(G[7] == 0.0)

@@ -169,6 +169,16 @@ int gmm_build_posting_lists(gmm_ctx* ctx, const int32_t* idx, const float* resp,
 int gmm_kmeans_step(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const float* centroids,
                     int32_t* assign, int32_t* work, float* centroids_out, int64_t* counts, double* inertia);
 
+/* Per-point log-density under the mixture, log p(x_i) = log sum_k pi_k N(x_i | mu_k, diag var_k) (Section 2; the
+ * stable log-sum-exp of Section 3.2, whose per-point value Algorithm 1 keeps on chip): the quantity a kernel density
+ * estimate evaluates, which the paper's Discussion (Section 6) names as another user of the fused pattern.
+ *   X [N x D], pi [K], mu [K x D], var [K x D]: device fp32, as for gmm_em_step.
+ *   logp [N] fp32, device out (natural logarithm);  loglik (host out, may be NULL): their sum in float64.
+ * Runs the log-sum-exp kernel of the FP32 path at every shape (exact direct-difference logits): a per-point value has no
+ * averaging over points to absorb the tensor path's approximate logits.  Errors as gmm_em_step.  Synchronises the stream. */
+int gmm_score_samples(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const float* pi, const float* mu,
+                      const float* var, float* logp, double* loglik);
+
 /* Fisher-vector encoding of G groups of points under a fixed mixture: the per-group use of the fused pattern (log-sum-exp
  * over the K weighted Gaussian terms, then responsibility-weighted statistics) that the paper's Discussion (Section 6)
  * names.  The paper prints no formula; the standard definition is used.  For a group of T points with responsibilities

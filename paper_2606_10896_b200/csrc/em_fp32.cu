@@ -666,6 +666,17 @@ cudaError_t launch_lse_fp32(cudaStream_t s, const float* X, int64_t n, int D, in
     return cudaGetLastError();
 }
 
+// Per-point log-density output of gmm_score_samples: log Z (natural log) from the base-2 values lse_kernel left.
+static __global__ void logz_out_kernel(const double* __restrict__ logZ2, int64_t n, float* __restrict__ out) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) out[i] = (float)(logZ2[i] * 0.69314718055994530942);
+}
+
+cudaError_t launch_logz_out_fp32(cudaStream_t s, const double* logZ2, int64_t n, float* out) {
+    logz_out_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(logZ2, n, out);
+    return cudaGetLastError();
+}
+
 template <int M, typename ACC>
 static cudaError_t launch_topm_t(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu,
                                  const float* w2, const double* c2d, const float* g, int m, int32_t* idx, float* resp,

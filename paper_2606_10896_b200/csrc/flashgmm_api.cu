@@ -868,6 +868,37 @@ int gmm_kmeans_step(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const
     return GMM_OK;
 }
 
+int gmm_score_samples(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const float* pi, const float* mu,
+                      const float* var, float* logp, double* loglik) {
+    CHECK(check_shape(ctx, N, D, K));
+    CHECK(check_ptr(ctx, X, 4, "X"));
+    CHECK(check_ptr(ctx, pi, 4, "pi"));
+    CHECK(check_ptr(ctx, mu, 4, "mu"));
+    CHECK(check_ptr(ctx, var, 4, "var"));
+    CHECK(check_ptr(ctx, logp, 4, "logp"));
+    DeviceGuard guard(ctx->device);
+    CHECK(ensure_scratch(ctx, D, K));
+    CU(cudaMemsetAsync(&ctx->result()->status, 0, sizeof(int), ctx->stream));
+    KL(launch_prepare_fp32(ctx->stream, D, K, pi, mu, var, ctx->w2(), ctx->c2(), ctx->c2d(), ctx->center(), &ctx->result()->status));
+    if ((size_t)K * D > ((size_t)1 << 12)) ctx->launches++;
+    CU(cudaMemsetAsync(&ctx->result()->ll[0], 0, 8, ctx->stream));
+    // the log-sum-exp kernel of the FP32 path, one super-tile at a time; its per-point values go out instead of into an M-step
+    for (int64_t off = 0; off < N; off += SUPER_TILE) {
+        const int64_t cnt = (N - off < SUPER_TILE) ? (N - off) : SUPER_TILE;
+        CHECK(prof_begin(ctx));
+        KL(launch_lse_fp32(ctx->stream, X + off * D, cnt, D, K, mu, ctx->w2(), ctx->c2d(), ctx->center(), ctx->logZ2(), ctx->llpart()));
+        CHECK(prof_end(ctx));
+        KL(launch_logz_out_fp32(ctx->stream, ctx->logZ2(), cnt, logp + off));
+        KL(launch_reduce_ll(ctx->stream, ctx->llpart(), (cnt + FP32_TILE_P - 1) / FP32_TILE_P, &ctx->result()->ll[0], true));
+    }
+    ctx->last_path = GMM_PATH_FP32;
+    double total = 0.0;
+    const int rc = read_result(ctx, 0, &total);
+    if (rc != GMM_OK) return rc;
+    if (loglik) *loglik = total;
+    return GMM_OK;
+}
+
 int gmm_fisher_vectors(gmm_ctx* ctx, const float* X, int64_t N, const int64_t* offsets, int G, int D, int K,
                        const float* pi, const float* mu, const float* var, float* fv, double* loglik) {
     CHECK(check_shape(ctx, N, D, K));

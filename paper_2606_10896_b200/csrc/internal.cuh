@@ -37,6 +37,8 @@ cudaError_t launch_center_fp32(cudaStream_t s, int D, int K, const float* mu, fl
 // gives the same mathematics, a centre near the data keeps the fp32 rounding small)
 cudaError_t launch_lse_fp32(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu,
                             const float* w2, const double* c2d, const float* g, double* logZ2, double* llpart);
+// out[i] = ln 2 * logZ2[i]: the per-point log-density in natural units, fp32
+cudaError_t launch_logz_out_fp32(cudaStream_t s, const double* logZ2, int64_t n, float* out);
 cudaError_t launch_mstep_fp32(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu,
                               const float* w2, const double* c2d, const float* g, const double* logZ2, float* partials,
                               const Fp32Plan& plan);

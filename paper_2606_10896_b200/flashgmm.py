@@ -57,6 +57,9 @@ EXPORTS = {
     "gmm_kmeans_step": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_int, ctypes.c_void_p,
                                        ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                        ctypes.POINTER(ctypes.c_double)]),
+    "gmm_score_samples": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_int,
+                                         ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                         ctypes.POINTER(ctypes.c_double)]),
     "gmm_fisher_vectors": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p, ctypes.c_int,
                                           ctypes.c_int, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                           ctypes.c_void_p, ctypes.POINTER(ctypes.c_double)]),
@@ -307,6 +310,18 @@ class Context:
                                          ctypes.byref(total), ctypes.byref(mean))
         self._check(rc)
         return offsets, items, int(total.value), float(mean.value)
+
+    def gmm_score_samples(self, X, pi, mu, var, out=None):
+        """Per-point log-density: (logp float32 [N], their float64 sum)."""
+        N, D = X.shape
+        K = mu.shape[0]
+        logp = out if out is not None else torch.empty(N, dtype=torch.float32, device=X.device)
+        ll = ctypes.c_double(0.0)
+        rc = lib.gmm_score_samples(self._h, _dev(X, torch.float32, (N, D), "X"), N, D, K, _dev(pi, torch.float32, (K,), "pi"),
+                                   _dev(mu, torch.float32, (K, D), "mu"), _dev(var, torch.float32, (K, D), "var"),
+                                   _dev(logp, torch.float32, (N,), "logp"), ctypes.byref(ll))
+        self._check(rc)
+        return logp, float(ll.value)
 
     def gmm_fisher_vectors(self, X, offsets, pi, mu, var, out=None):
         """Fisher vectors of the groups of consecutive rows given by ``offsets`` (host int64 [G + 1]):

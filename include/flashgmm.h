@@ -194,8 +194,12 @@ int gmm_score_samples(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, con
  *   fv [G x 2 x K x D] fp32, device out: per group the means part [K x D], then the standard-deviations part [K x D].
  *   No power or L2 normalisation is applied.
  *   loglik (host out, may be NULL): the total log-likelihood of all the groups' points.
- * Accuracy: that of the statistics (about 1e-6 of the data scale, relative to N_k), so a coordinate is exact to about
- * 1e-5 (1 + |G|) when |mu| / sigma is moderate; data far from the origin in units of sigma should be centred first.
+ * On the tensor-core path several groups share a launch (each group of CTAs accumulates one of them); groups too large
+ * for that are accumulated one at a time.  The result of a group does not depend on which other groups the call holds.
+ * Accuracy: a coordinate is a difference of the raw moments (N_k, S1, S2), which carry about 4e-6 relative error, so
+ * with A_k = N_k / (T sqrt(pi_k)) (at most about 1 for a group that resembles the mixture, up to 1 / sqrt(pi_k) for a
+ * group that sits on one light component) the error is about 2e-5 (1 + max|G|) + A_k (1e-3 + 4e-5 (1 + mu^2 / var));
+ * data far from the origin in units of sigma should be centred first.
  * Errors as gmm_em_step; GMM_EINVAL for offsets out of order or out of range.  Synchronises the stream. */
 int gmm_fisher_vectors(gmm_ctx* ctx, const float* X, int64_t N, const int64_t* offsets, int G, int D, int K,
                        const float* pi, const float* mu, const float* var, float* fv, double* loglik);

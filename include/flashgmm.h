@@ -195,7 +195,7 @@ int gmm_score_samples(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, con
  *   No power or L2 normalisation is applied.
  *   loglik (host out, may be NULL): the total log-likelihood of all the groups' points.
  * On the tensor-core path several groups share a launch (each group of CTAs accumulates one of them); groups too large
- * for that are accumulated one at a time.  The result of a group does not depend on which other groups the call holds.
+ * for that are accumulated one at a time.
  * Accuracy: a coordinate is a difference of the raw moments (N_k, S1, S2), which carry about 4e-6 relative error, so
  * with A_k = N_k / (T sqrt(pi_k)) (at most about 1 for a group that resembles the mixture, up to 1 / sqrt(pi_k) for a
  * group that sits on one light component) the error is about 2e-5 (1 + max|G|) + A_k (1e-3 + 4e-5 (1 + mu^2 / var));

@@ -467,6 +467,7 @@ struct RefineArgs {
     float e_launch; int n_ill;
     int32_t* unc_rows; int* unc_count;      // rows left to the exact kernel (row + row_offset), and their number
     int row_offset;                         // position of this piece inside the window of pieces that share the list
+    bool index_only;                        // the caller uses the indices alone: no demand on the accuracy of the log-sum-exp
 };
 
 // One point, the whole warp: exact evaluation of what matters (see assign_refine_kernel).  Lane q < LIST holds the q-th
@@ -594,7 +595,7 @@ __device__ __forceinline__ void refine_point(const RefineArgs& g, const TcIllCac
         if (Si > 0.f) ex += Si * fast_ex2(Mi - M);
         S = (s0 * fast_ex2(m0 - M) + s1 * fast_ex2(m1 - M) - ap) + ex;
         if (!(S > 0.f) || !(S < CUDART_INF_F)) certain = false;
-        else if (evaluated > 0 && !(S - ex <= 0.1f * S)) certain = false;
+        else if (!g.index_only && evaluated > 0 && !(S - ex <= 0.1f * S)) certain = false;
     }
     if (certain) {
         // lane j writes output j: from the exact list, then from the unevaluated candidates
@@ -628,11 +629,12 @@ __global__ void __launch_bounds__(256)
 assign_refine_kernel(const float* __restrict__ rec, const float* __restrict__ X, int64_t n, int D, int K,
                      const float* __restrict__ mu, const float* __restrict__ w2, const float* __restrict__ c2,
                      const int* __restrict__ flags, const TcIllCache* __restrict__ ill_cache, int m, int32_t* __restrict__ idx_out,
-                     float* __restrict__ resp_out, int32_t* __restrict__ unc_rows, int* __restrict__ unc_count, int row_offset) {
+                     float* __restrict__ resp_out, int32_t* __restrict__ unc_rows, int* __restrict__ unc_count, int row_offset,
+                     int index_only) {
     if (flags[3] != 0) return;
     constexpr int RECW = assign_recw(LIST);
     RefineArgs g;
-    g.unc_rows = unc_rows; g.unc_count = unc_count; g.row_offset = row_offset;
+    g.unc_rows = unc_rows; g.unc_count = unc_count; g.row_offset = row_offset; g.index_only = index_only != 0;
     g.X = X; g.n = n; g.D = D; g.K = K; g.mu = mu; g.w2 = w2; g.c2 = c2; g.m = m; g.idx_out = idx_out; g.resp_out = resp_out;
     g.e_launch = __int_as_float(flags[1]);          // error bound of the approximate logits from the parameters
     g.n_ill = flags[2];                             // ill-conditioned components (<= TC_MAX_ILL): left out of the approximate pass
@@ -733,7 +735,7 @@ assign_refine_kernel(const float* __restrict__ rec, const float* __restrict__ X,
 template <int LIST>
 cudaError_t launch_assign_t(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu, const float* w2,
                             const float* c2, const TcBuffers& tb, float* rec, int32_t* unc_rows, int* unc_count, int row_offset, int m,
-                            int32_t* idx, float* resp, int* status) {
+                            int32_t* idx, float* resp, int* status, bool index_only) {
     const TcPlan pl = tc_plan(D, K, 148);
     AssignParams p;
     p.n = n; p.n_chunks = pl.CL; p.n_ks = pl.n_ks;
@@ -768,7 +770,7 @@ cudaError_t launch_assign_t(cudaStream_t s, const float* X, int64_t n, int D, in
     const int64_t warps_wanted = batches < (int64_t)sms * 64 ? batches : (int64_t)sms * 64;
     const unsigned rgrid = (unsigned)((warps_wanted + 7) / 8);
     assign_refine_kernel<LIST, (LIST <= 6 ? 4 : GMM_MAX_TOPM)><<<rgrid, 256, 0, s>>>(rec, X, n, D, K, mu, w2, c2, tb.flags, tb.ill_cache, m, idx,
-                                                                               resp, unc_rows, unc_count, row_offset);
+                                                                               resp, unc_rows, unc_count, row_offset, index_only ? 1 : 0);
     return cudaGetLastError();
 }
 
@@ -789,10 +791,14 @@ size_t assign_tc_record_bytes(int m) { return (size_t)2 * assign_recw(m <= 4 ? 6
 
 cudaError_t launch_assign_tc(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu, const float* w2,
                              const float* c2, const TcBuffers& tb, float* rec, int32_t* unc_rows, int* unc_count, int row_offset, int m,
-                             int32_t* idx, float* resp, int* status) {
+                             int32_t* idx, float* resp, int* status, bool index_only) {
     if (n < 1 || n > TC_YPOINTS || m < 1 || m > GMM_MAX_TOPM) return cudaErrorInvalidValue;
-    if (m <= 4) return launch_assign_t<6>(s, X, n, D, K, mu, w2, c2, tb, rec, unc_rows, unc_count, row_offset, m, idx, resp, status);
-    return launch_assign_t<10>(s, X, n, D, K, mu, w2, c2, tb, rec, unc_rows, unc_count, row_offset, m, idx, resp, status);
+    // A caller that wants the nearest component alone (the k-means step) needs two candidates and the best value left
+    // outside, and no accurate log-sum-exp: the selection keeps 3 values per thread instead of 6.
+    if (index_only && m == 1)
+        return launch_assign_t<3>(s, X, n, D, K, mu, w2, c2, tb, rec, unc_rows, unc_count, row_offset, m, idx, resp, status, true);
+    if (m <= 4) return launch_assign_t<6>(s, X, n, D, K, mu, w2, c2, tb, rec, unc_rows, unc_count, row_offset, m, idx, resp, status, false);
+    return launch_assign_t<10>(s, X, n, D, K, mu, w2, c2, tb, rec, unc_rows, unc_count, row_offset, m, idx, resp, status, false);
 }
 
 }  // namespace fg

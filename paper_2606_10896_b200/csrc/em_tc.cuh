@@ -99,7 +99,8 @@ size_t assign_tc_record_bytes(int m);
 // caller runs launch_topm_fp32 over them (gather mode).
 cudaError_t launch_assign_tc(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu, const float* w2,
                              const float* c2, const TcBuffers& tb, float* rec, int32_t* unc_rows, int* unc_count, int row_offset,
-                             int m, int32_t* idx, float* resp, int* status);
+                             int m, int32_t* idx, float* resp, int* status, bool index_only = false);
+// index_only (with m = 1): the caller uses idx alone; resp is then only approximate.
 cudaError_t launch_reduce_tc(cudaStream_t s, int D, int K, int Q, const TcBuffers& tb, double* Nk, double* S1,
                              double* S2, bool accumulate);
 

@@ -654,7 +654,7 @@ int grow_buffer(gmm_ctx* ctx, void** buf, size_t* have, size_t need, const char*
 
 namespace {
 int assign_topm_impl(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const float* pi, const float* mu,
-                     const float* var, int m, int32_t* idx, float* resp);
+                     const float* var, int m, int32_t* idx, float* resp, bool index_only = false);
 }
 
 int gmm_assign_topm(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const float* pi, const float* mu,
@@ -675,7 +675,7 @@ int gmm_assign_topm(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const
 namespace {
 // The assignment pass proper (arguments checked, scratch in place); also the nearest-centroid search of the k-means step.
 int assign_topm_impl(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const float* pi, const float* mu,
-                     const float* var, int m, int32_t* idx, float* resp) {
+                     const float* var, int m, int32_t* idx, float* resp, bool index_only) {
     CU(cudaMemsetAsync(&ctx->result()->status, 0, sizeof(int), ctx->stream));
     KL(launch_prepare_fp32(ctx->stream, D, K, pi, mu, var, ctx->w2(), ctx->c2(), ctx->c2d(), ctx->center(), &ctx->result()->status));
     if ((size_t)K * D > ((size_t)1 << 12)) ctx->launches++;      // but for tiny problems, the centre of the means is a launch of its own
@@ -712,7 +712,8 @@ int assign_topm_impl(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, cons
             CHECK(prof_begin(ctx));
             KL(launch_transform_tc(ctx->stream, X + off * D, cnt, D, tb));
             KL(launch_assign_tc(ctx->stream, X + off * D, cnt, D, K, mu, ctx->w2(), ctx->c2(), tb, reinterpret_cast<float*>(base),
-                                unc_rows, unc_count, (int)(off - win_start), m, idx + off * m, resp + off * m, &ctx->result()->status));
+                                unc_rows, unc_count, (int)(off - win_start), m, idx + off * m, resp + off * m, &ctx->result()->status,
+                                index_only));
             ctx->launches++;
             ++in_window;
             if (in_window == WINDOW || off + piece >= N) {
@@ -844,7 +845,7 @@ int gmm_kmeans_step(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const
         float* var_u = static_cast<float*>(ctx->km_unit);
         float* pi_u = var_u + KD;
         KL(launch_kmeans_unit_mixture(ctx->stream, D, K, pi_u, var_u));
-        CHECK(assign_topm_impl(ctx, X, N, D, K, pi_u, centroids, var_u, 1, assign, resp));
+        CHECK(assign_topm_impl(ctx, X, N, D, K, pi_u, centroids, var_u, 1, assign, resp, true));       // the indices alone are used
     } else {
         KL(launch_kmeans_unit_params(ctx->stream, D, K, ctx->w2(), ctx->c2d()));
         KL(launch_center_fp32(ctx->stream, D, K, centroids, ctx->center()));

@@ -127,6 +127,8 @@ int gmm_fit(gmm_ctx* ctx, const float* X, int64_t N, int D, int K,
  * clusters with the largest responsibilities, which the caller thresholds with tau = 1/K).
  *   idx [N x m] int32 and resp [N x m] float32, device outputs; per point descending by responsibility, ties to the
  *   smaller component index.  1 <= m <= min(K, GMM_MAX_TOPM).  Asynchronous on the stream.
+ *   resp may be NULL: the indices alone are computed (the hard assignment of Section 4.2 with m = 1); the tensor-core
+ *   path then needs no accurate log-sum-exp and, for m = 1, keeps half as many candidates per point.
  * Where the tensor-core path applies (the rule of gmm_em_step) the logits of all components come from the tensor cores
  * as a selection pass and the best few per point are recomputed exactly in fp32, so indices and values are those of the
  * FP32 kernels; a point whose selection is not certain within the error bound of the selection pass is evaluated

@@ -608,7 +608,7 @@ __device__ __forceinline__ void refine_point(const RefineArgs& g, const TcIllCac
         const int k = from_top ? top.index_at(lane) : ka;
         if (lane < m) {
             g.idx_out[row * m + lane] = k;
-            g.resp_out[row * m + lane] = __fdividef(fast_ex2(v - M), S);
+            if (g.resp_out) g.resp_out[row * m + lane] = __fdividef(fast_ex2(v - M), S);
         }
         return;
     }
@@ -706,7 +706,7 @@ assign_refine_kernel(const float* __restrict__ rec, const float* __restrict__ X,
             for (int j = 0; j < LIST; ++j) {
                 if (j < m) {
                     idx_out[row * m + j] = al.i[j];
-                    resp_out[row * m + j] = __fdividef(fast_ex2(al.a[j] - M), S);
+                    if (resp_out) resp_out[row * m + j] = __fdividef(fast_ex2(al.a[j] - M), S);
                 }
             }
 #ifdef FLASHGMM_DEBUG

@@ -276,7 +276,7 @@ __device__ __forceinline__ void lse_tile(unsigned char* smem_raw, int64_t blk, c
                     ci[best] = -1;
                 }
                 idx_out[out_row * m_out + j] = id;
-                resp_out[out_row * m_out + j] = r;
+                if (resp_out) resp_out[out_row * m_out + j] = r;
             }
         }
     }

@@ -665,11 +665,11 @@ int gmm_assign_topm(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const
     CHECK(check_ptr(ctx, mu, 4, "mu"));
     CHECK(check_ptr(ctx, var, 4, "var"));
     CHECK(check_ptr(ctx, idx, 4, "idx"));
-    CHECK(check_ptr(ctx, resp, 4, "resp"));
+    if (resp) CHECK(check_ptr(ctx, resp, 4, "resp"));
     if (m < 1 || m > K || m > GMM_MAX_TOPM) return fail(ctx, GMM_EINVAL, "m must be in [1, min(K, %d)] (got %d)", GMM_MAX_TOPM, m);
     DeviceGuard g(ctx->device);
     CHECK(ensure_scratch(ctx, D, K));
-    return assign_topm_impl(ctx, X, N, D, K, pi, mu, var, m, idx, resp);
+    return assign_topm_impl(ctx, X, N, D, K, pi, mu, var, m, idx, resp, resp == nullptr);
 }
 
 namespace {
@@ -712,7 +712,7 @@ int assign_topm_impl(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, cons
             CHECK(prof_begin(ctx));
             KL(launch_transform_tc(ctx->stream, X + off * D, cnt, D, tb));
             KL(launch_assign_tc(ctx->stream, X + off * D, cnt, D, K, mu, ctx->w2(), ctx->c2(), tb, reinterpret_cast<float*>(base),
-                                unc_rows, unc_count, (int)(off - win_start), m, idx + off * m, resp + off * m, &ctx->result()->status,
+                                unc_rows, unc_count, (int)(off - win_start), m, idx + off * m, resp ? resp + off * m : nullptr, &ctx->result()->status,
                                 index_only));
             ctx->launches++;
             ++in_window;
@@ -721,7 +721,7 @@ int assign_topm_impl(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, cons
                 // tile kernel.  (One launch per window: with a few hundred rows per piece a launch per piece is all latency.)
                 const int64_t win_rows = off + cnt - win_start;
                 KL(launch_topm_fp32(ctx->stream, X + win_start * D, win_rows, D, K, mu, ctx->w2(), ctx->c2d(), ctx->center(), m,
-                                    idx + win_start * m, resp + win_start * m, nullptr, unc_rows, unc_count));
+                                    idx + win_start * m, resp ? resp + win_start * m : nullptr, nullptr, unc_rows, unc_count));
                 in_window = 0;
             }
             CHECK(prof_end(ctx));
@@ -730,7 +730,7 @@ int assign_topm_impl(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, cons
     }
     for (int64_t off = 0; off < N; off += SUPER_TILE) {
         const int64_t cnt = (N - off < SUPER_TILE) ? (N - off) : SUPER_TILE;
-        KL(launch_topm_fp32(ctx->stream, X + off * D, cnt, D, K, mu, ctx->w2(), ctx->c2d(), ctx->center(), m, idx + off * m, resp + off * m, run_fp32_if));
+        KL(launch_topm_fp32(ctx->stream, X + off * D, cnt, D, K, mu, ctx->w2(), ctx->c2d(), ctx->center(), m, idx + off * m, resp ? resp + off * m : nullptr, run_fp32_if));
     }
     ctx->last_path = tensor ? GMM_PATH_TENSOR : GMM_PATH_FP32;
     return GMM_OK;

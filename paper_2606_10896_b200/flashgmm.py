@@ -278,15 +278,23 @@ class Context:
         self._check(rc)
         return trace[: done.value].copy(), done.value
 
-    def gmm_assign_topm(self, X, pi, mu, var, m, out=None):
-        """(idx int32 [N, m], resp float32 [N, m]) CUDA tensors; asynchronous on the context's stream."""
+    def gmm_assign_topm(self, X, pi, mu, var, m, out=None, indices_only=False):
+        """(idx int32 [N, m], resp float32 [N, m]) CUDA tensors; asynchronous on the context's stream.
+        indices_only: resp is not computed (returned as None; ``out`` is then (idx, None))."""
         N, D = X.shape
         K = pi.shape[0]
         if out is None:
             idx = torch.empty((N, m), dtype=torch.int32, device=X.device)
-            resp = torch.empty((N, m), dtype=torch.float32, device=X.device)
+            resp = None if indices_only else torch.empty((N, m), dtype=torch.float32, device=X.device)
         else:
             idx, resp = out
+        if resp is None:
+            rc = lib.gmm_assign_topm(self._h, _dev(X, torch.float32, (N, D), "X"), N, D, K,
+                                     _dev(pi, torch.float32, (K,), "pi"), _dev(mu, torch.float32, (K, D), "mu"),
+                                     _dev(var, torch.float32, (K, D), "var"), int(m),
+                                     _dev(idx, torch.int32, (N, m), "idx"), None)
+            self._check(rc)
+            return idx, None
         rc = lib.gmm_assign_topm(self._h, _dev(X, torch.float32, (N, D), "X"), N, D, K,
                                  _dev(pi, torch.float32, (K,), "pi"), _dev(mu, torch.float32, (K, D), "mu"),
                                  _dev(var, torch.float32, (K, D), "var"), int(m),

@@ -413,6 +413,35 @@ def test_topm_tensor_path_against_oracle(fg, ctx, N, D, K, m):
     _topm_tensor_vs_oracle(fg, ctx, X, pi, mu, var, m, f"tensor top-m N={N} D={D} K={K} m={m}")
 
 
+@pytest.mark.parametrize("N,D,K,m,path", [(3000, 128, 1024, 1, "tensor"), (2500, 64, 200, 4, "tensor"), (1100, 96, 4096, 1, "tensor"),
+                                          (2000, 100, 300, 8, "tensor"), (2000, 16, 8, 2, "fp32"), (900, 130, 70, 1, "fp32")])
+def test_topm_indices_only(fg, ctx, N, D, K, m, path):
+    """gmm_assign_topm without a responsibility array (the hard assignment of Section 4.2 for m = 1): the indices must be
+    those the oracle ranks first; the values used for the comparison are the oracle's own responsibilities at the GPU's
+    indices.  Also at the initial parameters of config 2, where posteriors are broad."""
+    cases = [_random_mixture(np.random.default_rng(N + D + K + m), N, D, K)]
+    if K == 1024:
+        spec = synth.CONFIGS[2].with_n(N)
+        Xc = synth.sample_host(spec)
+        cases.append((Xc,) + tuple(synth.init_params(Xc, spec)))
+    for X, pi, mu, var in cases:
+        ctx.gmm_set_path(fg.GMM_PATH_TENSOR if path == "tensor" else fg.GMM_PATH_FP32)
+        idx_r, resp_r, next_r = orc.topm(X, pi, mu, var, m)
+        idx_g, none = ctx.gmm_assign_topm(_t(X), _t(pi), _t(mu), _t(var), m, indices_only=True)
+        torch.cuda.synchronize()
+        assert none is None
+        idx_g = idx_g.cpu().numpy()
+        assert idx_g.min() >= 0 and idx_g.max() < K
+        R = orc.responsibilities(X, pi, mu, var)[0]
+        resp_at = np.take_along_axis(R, idx_g.astype(np.int64), axis=1)
+        assert_topm_matches(idx_g, resp_at, idx_r, resp_r, next_r, what=f"indices only N={N} D={D} K={K} m={m}")
+        # and the same indices as the call that also returns the values, except where those tie
+        idx_f, resp_f = ctx.gmm_assign_topm(_t(X), _t(pi), _t(mu), _t(var), m)
+        torch.cuda.synchronize()
+        differ = (idx_f.cpu().numpy() != idx_g).any(axis=1)
+        assert differ.mean() <= 0.01
+
+
 def test_topm_tensor_path_after_em_iterations(fg, ctx):
     spec = synth.CONFIGS[2].with_n(3000)
     X = synth.sample_host(spec)

@@ -41,7 +41,7 @@ def parse():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--path", default="auto", choices=["auto", "fp32", "tensor"])
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--fisher-points", type=int, default=0,
+    ap.add_argument("--fisher-points", type=int, default=10000,
                     help="also time gmm_fisher_vectors over the first (at most 2M) points of X in groups of this many "
                          "consecutive points (outside the timed region; reported as 'fisher_vectors'); 0 skips it")
     ap.add_argument("--assign-m", type=int, default=4,

@@ -45,7 +45,7 @@ def parse():
                     help="also time gmm_fisher_vectors over the first (at most 2M) points of X in groups of this many "
                          "consecutive points (outside the timed region; reported as 'fisher_vectors'); 0 skips it")
     ap.add_argument("--assign-m", type=int, default=4,
-                    help="also time gmm_assign_topm with this m on the same X (after the timed EM steps, outside their "
+                    help="also time gmm_assign_topm with this m (and the hard assignment: m = 1, indices only) on the same X (after the timed EM steps, outside their "
                          "timed region; reported as 'assign_topm'); 0 skips it")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
@@ -294,6 +294,17 @@ def main():
                   "path": "tensor" if ctx.gmm_last_path() == fg.GMM_PATH_TENSOR else "fp32",
                   "mean_top1_resp": float(resp[:, 0].mean().item())}
         del idx, resp
+        # the hard assignment (m = 1, indices only)
+        idx1 = torch.empty((N, 1), dtype=torch.int32, device=dev)
+        ctx.gmm_assign_topm(X, pi, mu, var, 1, out=(idx1, None))
+        torch.cuda.synchronize()
+        a0.record()
+        for _ in range(reps):
+            ctx.gmm_assign_topm(X, pi, mu, var, 1, out=(idx1, None))
+        a1.record()
+        torch.cuda.synchronize()
+        assign["hard_assignment_ms"] = a0.elapsed_time(a1) / reps
+        del idx1
 
     # ---- optional: Fisher vectors of groups of consecutive points of the same X, under the same parameters ----
     fisher = None

@@ -8,9 +8,9 @@ sigma / sqrt(2 pi)), the closed form for one component, the vanishing gradient a
 hand-computed two-point case.  The GPU path goes through the per-group sufficient statistics (N_k, S1, S2) instead, so
 it shares no formula with the oracle.
 
-Tolerance of the GPU comparison, per coordinate (k, d) of a group of T points, with A_k = N_k / (T sqrt(pi_k)) the factor
-by which the group's share of component k exceeds the component's weight (about sqrt(pi_k) <= 1 for a group that
-resembles the mixture, up to 1 / sqrt(pi_k) for a group that sits on one light component):
+Tolerance of the GPU comparison, per coordinate (k, d) of a group of T points, with A_k = N_k / (T sqrt(pi_k)), the
+group's share N_k / T of component k over the square root of the component's weight (about sqrt(pi_k) <= 1 for a group
+that resembles the mixture, up to 1 / sqrt(pi_k) for a group that sits on one light component):
 
     2e-5 (1 + max|G|)  +  A_k (0.5 e + 4e-5 (1 + mu_kd^2 / var_kd))
 

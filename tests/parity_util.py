@@ -44,34 +44,64 @@ def assert_stats_close(N, s, got, ref, what=""):
     assert e2 <= 1e-4 * s * s, f"{what}: S2/N_k off by {e2:.3e} > {1e-4 * s * s:.3e}"
 
 
-def assert_topm_matches(idx_g, resp_g, idx_r, resp_r, next_r, tie=1e-6, what=""):
-    """Index sets equal except for ties within `tie` in responsibility; values within 1e-5 absolute + 1e-4 relative."""
+def oracle_resp_at(orc, X, pi, mu, var, idx, chunk=2048):
+    """The oracle's responsibilities r_ik at the given indices idx [N, m] (float64 [N, m]), evaluated row block by
+    row block so that the full N x K matrix of a large case is never held."""
+    idx = np.asarray(idx).astype(np.int64)
+    out = np.empty(idx.shape, np.float64)
+    for lo in range(0, len(X), chunk):
+        R = orc.responsibilities(X[lo:lo + chunk], pi, mu, var)[0]
+        out[lo:lo + chunk] = np.take_along_axis(R, idx[lo:lo + chunk], axis=1)
+    return out
+
+
+def topm_disagreements(idx_g, resp_g, idx_r, resp_r, next_r, r_at_g, tie=1e-6, check_values=True):
+    """Number of points whose top-m result breaks the rule below (a list of the reasons comes with it).
+
+    The rule (ties within `tie` = 1e-6 in responsibility may resolve either way; everything is judged by the ORACLE's
+    responsibilities, never by the values the GPU reports):
+      * a GPU index outside the oracle's set is accepted iff the oracle's r at that index is within `tie` of the
+        oracle's m-th largest r;
+      * an oracle choice the GPU dropped (the m-th included) is accepted iff it is within `tie` of the oracle's
+        (m+1)-th largest r;
+      * every reported value agrees with the oracle's r at the same index to 1e-5 absolute + 1e-4 relative;
+      * the reported values descend up to the tie width.
+    r_at_g [N, m]: the oracle's r at the GPU's indices (oracle_resp_at)."""
     idx_g = np.asarray(idx_g)
-    resp_g = np.asarray(resp_g, np.float64)
+    r_at_g = np.asarray(r_at_g, np.float64)
     N, m = idx_r.shape
-    bad = 0
+    bad, why = 0, []
     for i in range(N):
+        reasons = []
         sg, sr = set(idx_g[i].tolist()), set(idx_r[i].tolist())
         if len(sg) != m:
-            raise AssertionError(f"{what}: point {i} has repeated indices {idx_g[i]}")
-        if sg != sr:
-            # every oracle choice that the GPU dropped must tie with the oracle's (m+1)-th value or the m-th value
-            thresh = resp_r[i, m - 1]
-            for k in sr - sg:
-                j = int(np.where(idx_r[i] == k)[0][0])
-                if resp_r[i, j] - next_r[i] > tie and resp_r[i, j] - thresh > tie:
-                    bad += 1
-            for k in sg - sr:
-                j = int(np.where(idx_g[i] == k)[0][0])
-                if abs(resp_g[i, j] - thresh) > tie + 1e-4 * thresh and thresh - resp_g[i, j] > tie:
-                    bad += 1
-        else:
-            ref_map = dict(zip(idx_r[i].tolist(), resp_r[i].tolist()))
-            for j in range(m):
-                r = ref_map[int(idx_g[i, j])]
-                if abs(resp_g[i, j] - r) > 1e-5 + 1e-4 * r:
-                    bad += 1
-        # descending order up to the tie width
-        if (np.diff(resp_g[i]) > tie + 1e-4 * resp_g[i, :-1]).any():
+            reasons.append(f"repeated indices {idx_g[i].tolist()}")
+        mth = resp_r[i, m - 1]
+        for k in sr - sg:
+            j = int(np.where(idx_r[i] == k)[0][0])
+            if resp_r[i, j] - next_r[i] > tie:
+                reasons.append(f"dropped oracle choice {k} (r={resp_r[i, j]:.3e}, (m+1)-th={next_r[i]:.3e})")
+        for j in range(m):
+            k = int(idx_g[i, j])
+            if k not in sr and mth - r_at_g[i, j] > tie:
+                reasons.append(f"extra index {k} (oracle r={r_at_g[i, j]:.3e}, m-th={mth:.3e})")
+        if check_values:
+            rg = np.asarray(resp_g[i], np.float64)
+            if (np.abs(rg - r_at_g[i]) > 1e-5 + 1e-4 * r_at_g[i]).any():
+                reasons.append(f"values {rg.tolist()} vs oracle {r_at_g[i].tolist()}")
+            if (np.diff(rg) > tie + 1e-4 * rg[:-1]).any():
+                reasons.append(f"values not descending {rg.tolist()}")
+        else:           # indices only: the oracle's values at the GPU's indices must descend
+            if (np.diff(r_at_g[i]) > tie).any():
+                reasons.append(f"indices not in descending order of the oracle's r {r_at_g[i].tolist()}")
+        if reasons:
             bad += 1
-    assert bad == 0, f"{what}: {bad} top-m disagreements beyond the tie rule"
+            if len(why) < 5:
+                why.append(f"point {i}: " + "; ".join(reasons))
+    return bad, why
+
+
+def assert_topm_matches(idx_g, resp_g, idx_r, resp_r, next_r, r_at_g, tie=1e-6, what="", check_values=True):
+    """See topm_disagreements."""
+    bad, why = topm_disagreements(idx_g, resp_g, idx_r, resp_r, next_r, r_at_g, tie, check_values)
+    assert bad == 0, f"{what}: {bad} top-m disagreements beyond the tie rule: " + " | ".join(why)

@@ -10,7 +10,7 @@ import torch
 
 from oracle import gmm_oracle as orc
 from paper_2606_10896_b200 import synth
-from tests.parity_util import assert_params_close, assert_stats_close, assert_topm_matches, data_scale
+from tests.parity_util import assert_params_close, assert_stats_close, assert_topm_matches, data_scale, oracle_resp_at
 
 pytestmark = pytest.mark.gpu
 
@@ -46,6 +46,16 @@ def _paths(fg, D, K):
 def _gpu_step(ctx, X_d, pi, mu, var):
     Nk, S1, S2, L = ctx.gmm_em_step(X_d, _t(pi), _t(mu), _t(var))
     return Nk.cpu().numpy(), S1.cpu().numpy(), S2.cpu().numpy(), L
+
+
+def _check_topm(X, pi, mu, var, m, idx_g, resp_g, what):
+    """The GPU's top-m rows against the oracle's under the tie rule of tests/parity_util.py; resp_g = None checks the
+    indices alone."""
+    idx_g = np.asarray(idx_g)
+    idx_r, resp_r, next_r = orc.topm(X, pi, mu, var, m)
+    r_at_g = oracle_resp_at(orc, X, pi, mu, var, idx_g)
+    assert idx_g.min() >= 0 and idx_g.max() < len(pi), f"{what}: index out of range"
+    assert_topm_matches(idx_g, resp_g, idx_r, resp_r, next_r, r_at_g, what=what, check_values=resp_g is not None)
 
 
 def _teacher_forced(fg, ctx, X, spec, iters, paths=None):
@@ -379,10 +389,9 @@ def test_topm_against_oracle(fg, ctx, cfg, n, m):
     pi0, mu0, var0 = synth.init_params(X, spec)
     fit = orc.fit(X, pi0, mu0, var0, 3, var_floor=spec.var_floor)
     p32, m32, v32 = (fit[k].astype(np.float32) for k in ("pi", "mu", "var"))
-    idx_r, resp_r, next_r = orc.topm(X, p32, m32, v32, m)
     idx_g, resp_g = ctx.gmm_assign_topm(_t(X), _t(p32), _t(m32), _t(v32), m)
     torch.cuda.synchronize()
-    assert_topm_matches(idx_g.cpu().numpy(), resp_g.cpu().numpy(), idx_r, resp_r, next_r, what=f"cfg {cfg} m {m}")
+    _check_topm(X, p32, m32, v32, m, idx_g.cpu().numpy(), resp_g.cpu().numpy(), f"cfg {cfg} m {m}")
 
 
 def _random_mixture(rng, N, D, K, spread=2.0):
@@ -395,11 +404,10 @@ def _random_mixture(rng, N, D, K, spread=2.0):
 
 def _topm_tensor_vs_oracle(fg, ctx, X, pi, mu, var, m, what, expect_path=None):
     ctx.gmm_set_path(fg.GMM_PATH_TENSOR)
-    idx_r, resp_r, next_r = orc.topm(X, pi, mu, var, m)
     idx_g, resp_g = ctx.gmm_assign_topm(_t(X), _t(pi), _t(mu), _t(var), m)
     torch.cuda.synchronize()
     assert ctx.gmm_last_path() == (expect_path or fg.GMM_PATH_TENSOR)
-    assert_topm_matches(idx_g.cpu().numpy(), resp_g.cpu().numpy(), idx_r, resp_r, next_r, what=what)
+    _check_topm(X, pi, mu, var, m, idx_g.cpu().numpy(), resp_g.cpu().numpy(), what)
 
 
 @pytest.mark.parametrize("N,D,K,m", [(1500, 128, 1024, 4), (777, 30, 100, 2), (2000, 100, 200, 8), (300, 9, 1000, 1),
@@ -426,15 +434,11 @@ def test_topm_indices_only(fg, ctx, N, D, K, m, path):
         cases.append((Xc,) + tuple(synth.init_params(Xc, spec)))
     for X, pi, mu, var in cases:
         ctx.gmm_set_path(fg.GMM_PATH_TENSOR if path == "tensor" else fg.GMM_PATH_FP32)
-        idx_r, resp_r, next_r = orc.topm(X, pi, mu, var, m)
         idx_g, none = ctx.gmm_assign_topm(_t(X), _t(pi), _t(mu), _t(var), m, indices_only=True)
         torch.cuda.synchronize()
         assert none is None
         idx_g = idx_g.cpu().numpy()
-        assert idx_g.min() >= 0 and idx_g.max() < K
-        R = orc.responsibilities(X, pi, mu, var)[0]
-        resp_at = np.take_along_axis(R, idx_g.astype(np.int64), axis=1)
-        assert_topm_matches(idx_g, resp_at, idx_r, resp_r, next_r, what=f"indices only N={N} D={D} K={K} m={m}")
+        _check_topm(X, pi, mu, var, m, idx_g, None, f"indices only N={N} D={D} K={K} m={m}")
         # and the same indices as the call that also returns the values, except where those tie
         idx_f, resp_f = ctx.gmm_assign_topm(_t(X), _t(pi), _t(mu), _t(var), m)
         torch.cuda.synchronize()
@@ -514,7 +518,6 @@ def test_data_far_from_the_origin(fg, ctx):
     mu = (mu + 300.0).astype(np.float32)
     s = data_scale(X)
     ref = orc.em_step(X, pi, mu, var)
-    idx_r, resp_r, next_r = orc.topm(X, pi, mu, var, 3)
     for path in _paths(fg, D, K):
         ctx.gmm_set_path(path)
         got = _gpu_step(ctx, _t(X), pi, mu, var)
@@ -522,7 +525,7 @@ def test_data_far_from_the_origin(fg, ctx):
         assert_stats_close(N, s, got[:3], ref[:3], f"path {path}, data far from the origin")
         idx_g, resp_g = ctx.gmm_assign_topm(_t(X), _t(pi), _t(mu), _t(var), 3)
         torch.cuda.synchronize()
-        assert_topm_matches(idx_g.cpu().numpy(), resp_g.cpu().numpy(), idx_r, resp_r, next_r, what=f"path {path}, far from the origin")
+        _check_topm(X, pi, mu, var, 3, idx_g.cpu().numpy(), resp_g.cpu().numpy(), f"path {path}, far from the origin")
 
 
 @pytest.mark.parametrize("N,D,K", [(3000, 3, 1), (7001, 3, 5), (2000, 8, 2)])
@@ -599,8 +602,8 @@ def _full_size_topm_check(fg, ctx, X, spec, pi0, mu0, var0, what, n_rows=3000):
     assert int(idx.min()) >= 0 and int(idx.max()) < spec.K
     rows = synth.subsample_rows(spec.N, n_rows, spec.seed + 17)
     rows_d = torch.as_tensor(rows, device=DEV)
-    idx_r, resp_r, next_r = orc.topm(X[rows_d].cpu().numpy(), pi.cpu().numpy(), mu.cpu().numpy(), var.cpu().numpy(), 4)
-    assert_topm_matches(idx[rows_d].cpu().numpy(), resp[rows_d].cpu().numpy(), idx_r, resp_r, next_r, what=what)
+    _check_topm(X[rows_d].cpu().numpy(), pi.cpu().numpy(), mu.cpu().numpy(), var.cpu().numpy(), 4,
+                idx[rows_d].cpu().numpy(), resp[rows_d].cpu().numpy(), what)
 
 
 def _column_sums(X):
@@ -688,9 +691,8 @@ def test_config5_shape_step_and_topm_on_subsample(fg, ctx):
     assert abs(got[3] - ref[3]) <= 1e-5 * abs(ref[3])
     assert_stats_close(len(rows), data_scale(Xsub), got[:3], ref[:3], "config 5 subsample")
     p1, m1, v1 = pi_d.cpu().numpy(), mu_d.cpu().numpy(), var_d.cpu().numpy()
-    idx_r, resp_r, next_r = orc.topm(Xsub, p1, m1, v1, 4)
-    assert_topm_matches(idx[rows_d].cpu().numpy(), resp[rows_d].cpu().numpy(), idx_r, resp_r, next_r,
-                        what="config 5 top-4 subsample")
+    _check_topm(Xsub, p1, m1, v1, 4, idx[rows_d].cpu().numpy(), resp[rows_d].cpu().numpy(),
+                "config 5 top-4 subsample")
 
 
 def test_isotropic_update_and_fit_match_the_papers_model(fg, ctx):

@@ -1,6 +1,7 @@
 """gmm_em_step_static -- the entry point for callers that cannot allocate device memory (hosts whose device heap
 belongs to another allocator, or that may not block on the driver's allocator) -- checked through the C ABI against
-gmm_em_step on the same inputs, twice in a row so that stale contents of the shared static scratch would show.
+the float64 oracle and against gmm_em_step on the same inputs, twice in a row so that stale contents of the shared
+static scratch would show.
 
 Collected last on purpose: a run that stops at the first failure has then already run every other test.
 """
@@ -8,6 +9,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import gmm_oracle as orc
 from paper_2606_10896_b200 import synth
 from tests.parity_util import assert_stats_close, data_scale
 
@@ -37,6 +39,7 @@ def test_static_scratch_entry_point_matches_em_step_twice_in_a_row():
             X_d, pi_d, mu_d, var_d = _t(X), _t(pi), _t(mu), _t(var)
             Nk_r, S1_r, S2_r, L_r = ctx.gmm_em_step(X_d, pi_d, mu_d, var_d)
             ref = (Nk_r.cpu().numpy(), S1_r.cpu().numpy(), S2_r.cpu().numpy())
+            Nk_o, S1_o, S2_o, L_o = orc.em_step(X, pi, mu, var)          # the float64 definition, same fp32 inputs
             out = (torch.full((K,), 7.0, dtype=torch.float64, device=DEV),
                    torch.full((K, D), -3.0, dtype=torch.float64, device=DEV),
                    torch.full((K, D), 5.0, dtype=torch.float64, device=DEV))
@@ -47,6 +50,8 @@ def test_static_scratch_entry_point_matches_em_step_twice_in_a_row():
                 assert abs(L - L_r) <= 1e-5 * abs(L_r), (call, L, L_r)
                 assert abs(got[0].sum() - N) <= 1e-5 * N
                 assert_stats_close(N, s, got, ref, f"static call {call} shape {(N, D, K)}")
+                assert abs(L - L_o) <= 1e-5 * abs(L_o), (call, L, L_o)
+                assert_stats_close(N, s, got, (Nk_o, S1_o, S2_o), f"static call {call} vs oracle, shape {(N, D, K)}")
                 if first is None:
                     first = (L, got)
                 else:       # same inputs, same launch configuration: the same bits

@@ -20,6 +20,9 @@
  *     gmm_last_error(ctx) gives a human-readable message.  Output arrays are unspecified after a failure.
  *   - Work is enqueued on the context's stream; a call that has a host output synchronises that stream before it
  *     returns, calls without host outputs (gmm_finalize, gmm_assign_topm) return with the work still in flight.
+ *     What device code finds wrong (invalid parameters, an expired wait) is recorded in a status word that stays set
+ *     until the host has reported it: for an asynchronous call that is the next synchronising call on the context, or
+ *     gmm_sync_status.
  *   - Results are deterministic: the same inputs give the same bits on every call (no floating-point atomics;
  *     per-CTA partial sums are added in a fixed order in float64).
  *   - A context is not thread-safe; use one per host thread.
@@ -39,7 +42,7 @@ extern "C" {
 #define GMM_EALIGN   -2   /* a pointer is not aligned for its element type */
 #define GMM_ENOMEM   -3   /* scratch allocation failed */
 #define GMM_ECUDA    -4   /* a CUDA call failed; message in gmm_last_error */
-#define GMM_ENUMERIC -5   /* var <= 0, pi < 0, non-finite parameter, or non-finite log-likelihood */
+#define GMM_ENUMERIC -5   /* var <= 0, pi < 0, non-finite parameter, non-finite value in X, or non-finite log-likelihood */
 #define GMM_ETIMEOUT -6   /* a bounded device-side wait expired; results invalid */
 #define GMM_EUNSUPPORTED -7 /* the requested kernel path cannot run this shape */
 
@@ -117,7 +120,9 @@ int gmm_set_covariance(gmm_ctx* ctx, int covariance);
  * repeatedly).  pi/mu/var: device, in = initial parameters, out = fitted.  loglik_trace: host [iters];
  * trace[t] is the log-likelihood under the parameters ENTERING iteration t.  tol > 0 stops after iteration t >= 1
  * when |L_t - L_{t-1}| <= tol * |L_t|; tol = 0 runs all iterations.  iters_done (host, may be NULL) receives the
- * number of iterations run.  Synchronises the stream. */
+ * number of iterations run.  If an iteration fails (GMM_ENUMERIC: invalid parameters or non-finite data; GMM_ETIMEOUT),
+ * its parameter update is not applied: pi, mu, var hold the parameters that entered the failed iteration.
+ * Synchronises the stream. */
 int gmm_fit(gmm_ctx* ctx, const float* X, int64_t N, int D, int K,
             float* pi, float* mu, float* var,
             int iters, float var_floor, double tol,
@@ -150,14 +155,14 @@ int gmm_assign_topm(gmm_ctx* ctx, const float* X, int64_t N, int D, int K,
  *   offsets [K + 1] int64, device out: list k holds items[offsets[k] .. offsets[k+1]).
  *   items  int32, device out, capacity >= N * max_lists entries: vector indices, ascending inside every list.
  *   total (host out, may be NULL): offsets[K];  mean_lists (host out, may be NULL): total / N, the paper's average
- *   number of posting lists per vector (Section 5, multi-assignment analysis).
+ *   number of posting lists per vector (Section 4.6, multi-assignment analysis).
  * Deterministic (no atomics on the output); scratch O(K), independent of N.  Limits: N < 2^31, K <= 8192 (otherwise
  * GMM_EUNSUPPORTED).  Synchronises the stream. */
 int gmm_build_posting_lists(gmm_ctx* ctx, const int32_t* idx, const float* resp, int64_t N, int m, int K,
                             float tau, int max_lists, int64_t* offsets, int32_t* items,
                             int64_t* total, double* mean_lists);
 
-/* One Lloyd (k-means) iteration, the warm start the paper runs before its EM iterations (Section 5, experimental setup:
+/* One Lloyd (k-means) iteration, the warm start the paper runs before its EM iterations (Section 4.4, experimental setup, and the warm-start appendix:
  * 10 iterations of k-means, then Flash-GMM).  Assignment: every point goes to the centroid at the smallest squared
  * Euclidean distance (direct differences in fp32; ties to the smaller index).  Update: a centroid becomes the mean of its
  * points (float64 sums in a fixed order); a centroid without points keeps its position.
@@ -229,6 +234,17 @@ int gmm_fisher_vectors(gmm_ctx* ctx, const float* X, int64_t N, const int64_t* o
 int gmm_em_step_static(int device, void* cuda_stream, const float* X, int64_t N, int D, int K,
                        const float* pi, const float* mu, const float* var,
                        double* Nk, double* S1, double* S2, double* loglik);
+
+/* Waits for the context's stream and reports what device code recorded since the last report: GMM_OK, or the error of
+ * an earlier asynchronous call (GMM_ENUMERIC for var <= 0, pi < 0 or non-finite parameters given to gmm_assign_topm;
+ * GMM_ETIMEOUT).  The outputs of that call are then invalid.  Reporting clears the record. */
+int gmm_sync_status(gmm_ctx* ctx);
+
+/* Diagnostics of the most recent parameter update on this context (gmm_finalize, gmm_finalize_isotropic, or the last
+ * iteration of gmm_fit): how many variance entries were raised to var_floor, and how many components were left
+ * unchanged because N_k < 1e-12.  (The paper has neither rule; both can break the monotone growth of the
+ * log-likelihood, so a caller watching the trace wants to know.)  Either output may be NULL.  Synchronises the stream. */
+int gmm_update_counts(gmm_ctx* ctx, int64_t* floored_variances, int64_t* empty_components);
 
 /* Bytes of device scratch a context in GMM_PATH_AUTO holds for shape (D, K); independent of N.  Where the tensor
  * path runs (see gmm_auto_path) this includes 512 MiB for the fp16 planes of one launch-sized piece of the data;

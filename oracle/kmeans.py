@@ -1,4 +1,4 @@
-"""CPU oracle of one Lloyd (k-means) iteration, the warm start the paper uses before its EM iterations (Section 5,
+"""CPU oracle of one Lloyd (k-means) iteration, the warm start the paper uses before its EM iterations (Section 4.4,
 experimental setup: 10 iterations of k-means, then Flash-GMM).
 
 TEST INFRASTRUCTURE ONLY: the tests call this; the product package never imports it.  Plain numpy in float64, written

@@ -3,9 +3,9 @@
 // Phase 1 (lse_kernel): for a tile of 64 points sweep all K components in blocks of 64, keep the running
 //   (max, sum) of the online log-sum-exp per point on chip, write log Z_i (paper Algorithm 1, Step 1).
 // Phase 2 (mstep_kernel): a CTA owns 64 components (and a 128-wide slice of D); for each of its point tiles it
-//   recomputes log z_ik, forms r_ik = exp(log z_ik - log Z_i) in shared memory and accumulates N_k, S1, S2 in
-//   registers across ALL its tiles (Algorithm 1, Step 2) -- the accumulators leave the SM once, as a per-CTA
-//   partial; there are no atomics.
+//   recomputes log z_ik, forms r_ik = exp(log z_ik - log Z_i) in shared memory and accumulates N_k and the CENTRED
+//   sums of r (x - g), r (x - g)^2 in registers across ALL its tiles (Algorithm 1, Step 2) -- the accumulators leave
+//   the SM once, as a per-CTA partial; there are no atomics.  The reduction shifts them back to S1, S2 in float64.
 // The arithmetic is in the log2 domain: w2 = (log2 e / 2) / var, c2 = log2 e * (log pi - 1/2 sum_d log(2 pi var)),
 // log2 z = c2 - sum_d w2 (x - mu)^2, so the exponential is a bare ex2.  A term w2 (x - mu)^2 is formed as t^2 with
 // t = (x - g) sqrt(w2) - (mu - g) sqrt(w2): one FMA for t (the second product is prepared when the tile is staged) and
@@ -368,7 +368,9 @@ mstep_kernel(const float* __restrict__ X, int64_t n, int D, int K, const float* 
             const int e = tid + j * NTHREADS, r = e >> 7, c = e & 127;
             const int64_t row = row0 + r;
             const int d = dz0 + c;
-            xm[r * LDX + c] = (row < n && d < D) ? __ldg(X + row * D + d) : 0.f;
+            // centred: the sums are taken of x - g and (x - g)^2 (the reduction shifts them back in float64), so that
+            // fp32 accumulation errors scale with the data's spread, not with its distance from the origin
+            xm[r * LDX + c] = (row < n && d < D) ? __ldg(X + row * D + d) - (g ? __ldg(g + d) : 0.f) : 0.f;
         }
         __syncthreads();
         if (tid < TC) {
@@ -497,7 +499,7 @@ mstep_wide_kernel(const float* __restrict__ X, int64_t n, int D, int K, const fl
                     const int e = tid + j * NTHREADS, r = e >> 7, c = e & 127;
                     const int64_t row = row0 + r;
                     const int d = dz0 + c;
-                    xm[r * LDX + c] = (row < n && d < D) ? __ldg(X + row * D + d) : 0.f;
+                    xm[r * LDX + c] = (row < n && d < D) ? __ldg(X + row * D + d) - (g ? __ldg(g + d) : 0.f) : 0.f;      // centred
                 }
                 __syncthreads();
                 const float* r_s = r_all + w * TP * LDR;

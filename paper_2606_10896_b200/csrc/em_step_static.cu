@@ -127,7 +127,7 @@ extern "C" int gmm_em_step_static(int device, void* cuda_stream, const float* X,
         SCU(launch_lse_fp32(s, Xs, cnt, D, K, mu, w2, c2d, center, logZ2, llpart));
         SCU(launch_mstep_fp32(s, Xs, cnt, D, K, mu, w2, c2d, center, logZ2, partials, plan));
         SCU(launch_reduce_ll(s, llpart, (cnt + FP32_TILE_P - 1) / FP32_TILE_P, &res->ll, true));
-        SCU(launch_reduce_partials(s, D, K, plan.splits, partials, Nk, S1, S2, true));
+        SCU(launch_reduce_partials(s, D, K, plan.splits, partials, center, Nk, S1, S2, true));
     }
     StaticResult h;
     SCU(cudaMemcpyAsync(&h, res, sizeof(StaticResult), cudaMemcpyDeviceToHost, s));

@@ -1069,14 +1069,16 @@ __device__ __forceinline__ void tc_load_unit(const float* __restrict__ X, int64_
 }
 
 __device__ __forceinline__ void tc_store_unit(const float (&x)[8], bool valid, const float* __restrict__ sd,
-                                              const float* __restrict__ kap, int64_t u, unsigned char* __restrict__ yhi,
-                                              unsigned char* __restrict__ ylo) {
+                                              const float* __restrict__ kap, const float* __restrict__ gd, int64_t u,
+                                              unsigned char* __restrict__ yhi, unsigned char* __restrict__ ylo) {
     const int64_t row = u >> 4;
     const int ks = (int)(u & 15), d0 = ks * 8;
     uint32_t xh[4], xl[4], qh[4], ql[4];
 #pragma unroll
     for (int j = 0; j < 8; j += 2) {
-        float u0 = x[j] * __ldg(sd + d0 + j), u1 = x[j + 1] * __ldg(sd + d0 + j + 1);
+        // centred and scaled: u = s_d (x - g_d)  (padded dimensions: s = 1, g = 0, x = 0)
+        float u0 = (x[j] - __ldg(gd + d0 + j)) * __ldg(sd + d0 + j), u1 = (x[j + 1] - __ldg(gd + d0 + j + 1)) * __ldg(sd + d0 + j + 1);
+        if (!valid) { u0 = 0.f; u1 = 0.f; }
         u0 = fminf(fmaxf(u0, -240.f), 240.f);
         u1 = fminf(fmaxf(u1, -240.f), 240.f);
         float q0 = fmaf(u0, u0, __ldg(kap + d0 + j)), q1 = fmaf(u1, u1, __ldg(kap + d0 + j + 1));
@@ -1102,18 +1104,25 @@ __device__ __forceinline__ void tc_store_unit(const float (&x)[8], bool valid, c
 
 __global__ void __launch_bounds__(256) tc_transform_kernel(const float* __restrict__ X, int64_t n, int64_t rows_padded, int D,
                                                            const float* __restrict__ sd, const float* __restrict__ kap,
-                                                           unsigned char* __restrict__ yhi, unsigned char* __restrict__ ylo) {
+                                                           const float* __restrict__ gd,
+                                                           unsigned char* __restrict__ yhi, unsigned char* __restrict__ ylo,
+                                                           int* __restrict__ status) {
     const bool vec_ok = (D % 4 == 0) && ((reinterpret_cast<uintptr_t>(X) & 15) == 0);
     const int64_t units = rows_padded * 16;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    bool bad = false;
     // two units per step, both loads issued before the first store: twice the bytes in flight per thread
     for (int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; u < units; u += 2 * stride) {
         float xa[8], xb[8];
         tc_load_unit(X, n, D, vec_ok, u, units, xa);
         tc_load_unit(X, n, D, vec_ok, u + stride, units, xb);
-        tc_store_unit(xa, (u >> 4) < n, sd, kap, u, yhi, ylo);
-        if (u + stride < units) tc_store_unit(xb, ((u + stride) >> 4) < n, sd, kap, u + stride, yhi, ylo);
+        // (the planes clamp every coordinate to a finite range, so a NaN or an infinity in X has to be caught here)
+#pragma unroll
+        for (int j = 0; j < 8; ++j) bad |= !(fabsf(xa[j]) <= 3.0e38f) || !(fabsf(xb[j]) <= 3.0e38f);
+        tc_store_unit(xa, (u >> 4) < n, sd, kap, gd, u, yhi, ylo);
+        if (u + stride < units) tc_store_unit(xb, ((u + stride) >> 4) < n, sd, kap, gd, u + stride, yhi, ylo);
     }
+    if (bad) atomicOr(status, ST_BAD_X);
 }
 
 // The same planes for a grouped launch: row r of the planes belongs to tile t = r / BN and holds point
@@ -1122,9 +1131,12 @@ __global__ void __launch_bounds__(256) tc_transform_grouped_kernel(const float* 
                                                                    const int* __restrict__ tile_valid,
                                                                    const int64_t* __restrict__ tile_src,
                                                                    const float* __restrict__ sd, const float* __restrict__ kap,
-                                                                   unsigned char* __restrict__ yhi, unsigned char* __restrict__ ylo) {
+                                                                   const float* __restrict__ gd,
+                                                                   unsigned char* __restrict__ yhi, unsigned char* __restrict__ ylo,
+                                                                   int* __restrict__ status) {
     const int64_t units = rows * 16;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    bool bad = false;
     for (int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; u < units; u += stride) {
         const int64_t row = u >> 4;
         const int64_t t = row / BN;
@@ -1134,14 +1146,19 @@ __global__ void __launch_bounds__(256) tc_transform_grouped_kernel(const float* 
         const int d0 = (int)(u & 15) * 8;
         float x[8];
 #pragma unroll
-        for (int q = 0; q < 8; ++q) x[q] = (valid && d0 + q < D) ? __ldg(xr + d0 + q) : 0.f;
-        tc_store_unit(x, valid, sd, kap, u, yhi, ylo);
+        for (int q = 0; q < 8; ++q) {
+            x[q] = (valid && d0 + q < D) ? __ldg(xr + d0 + q) : 0.f;
+            bad |= !(fabsf(x[q]) <= 3.0e38f);
+        }
+        tc_store_unit(x, valid, sd, kap, gd, u, yhi, ylo);
     }
+    if (bad) atomicOr(status, ST_BAD_X);
 }
 
 // ---------------------------------------------------------------------------------------------------------------
 // Parameter preparation for the tensor path (float64 arithmetic, K*D elements: negligible)
 
+// (All means below are taken about the per-dimension centre g_d, see the kernel.)
 // s_d = 2^-round(log2 rms_d) with rms_d^2 = sum_k pi_k (mu_kd^2 + var_kd): brings every dimension to O(1) so that the
 // fp16 splits keep their precision whatever the data's units.  kap_d = s_d^2 sum_k pi_k mu_kd^2: the squares enter the
 // contraction as (s x)^2 + kap_d, which turns the monotonically growing partial sums sum_d w (mu x - x^2 / 2) ~ sum_d w mu^2 / 2
@@ -1149,20 +1166,47 @@ __global__ void __launch_bounds__(256) tc_transform_grouped_kernel(const float* 
 // in the tensor core.  The constant is given back exactly through c_k (E-step) and kap_d N_k (M-step).
 __global__ void __launch_bounds__(128) tc_scale_kernel(int D, int K, const float* __restrict__ pi, const float* __restrict__ mu,
                                                        const float* __restrict__ var, float* __restrict__ sd,
-                                                       float* __restrict__ kap) {
-    // one block per dimension (padded to 128); threads stride over the components, fixed-shape tree reduction
+                                                       float* __restrict__ kap, float* __restrict__ gd) {
+    // one block per dimension (padded to 128); threads stride over the components, fixed-shape tree reductions.
+    // First the centre g_d = sum_k pi_k mu_kd / sum_k pi_k: points and means enter every product as x - g, mu - g, so that
+    // data far from the origin (in units of its spread) costs the fp16 splits and the fp32 accumulators no precision; the
+    // statistics are shifted back in float64 by the reduction.
     const int d = blockIdx.x, t = threadIdx.x;
     __shared__ double r_acc[128], r_m[128], r_w[128];
-    double acc = 0.0, accm = 0.0, wsum = 0.0;
+    __shared__ double g_s;
+    double accg = 0.0, wsum = 0.0;
     if (d < D) {
         for (int k = t; k < K; k += 128) {
             const double w = (double)pi[k];
-            const double m = (double)mu[(size_t)k * D + d];
+            accg += w * (double)mu[(size_t)k * D + d];
+            wsum += w;
+        }
+    }
+    r_acc[t] = accg; r_w[t] = wsum;
+    __syncthreads();
+    for (int o = 64; o > 0; o >>= 1) {
+        if (t < o) { r_acc[t] += r_acc[t + o]; r_w[t] += r_w[t + o]; }
+        __syncthreads();
+    }
+    if (t == 0) {
+        double g = (r_w[0] > 0.0) ? r_acc[0] / r_w[0] : 0.0;
+        const float gf = (float)g;                       // the kernels subtract the fp32 value: use exactly that one
+        g_s = (d < D && isfinite(gf)) ? (double)gf : 0.0;
+    }
+    __syncthreads();
+    const double g = g_s;
+    double acc = 0.0, accm = 0.0;
+    wsum = 0.0;
+    if (d < D) {
+        for (int k = t; k < K; k += 128) {
+            const double w = (double)pi[k];
+            const double m = (double)mu[(size_t)k * D + d] - g;
             acc += w * (m * m + (double)var[(size_t)k * D + d]);
             accm += w * m * m;
             wsum += w;
         }
     }
+    __syncthreads();
     r_acc[t] = acc; r_m[t] = accm; r_w[t] = wsum;
     __syncthreads();
     for (int o = 64; o > 0; o >>= 1) {
@@ -1176,10 +1220,11 @@ __global__ void __launch_bounds__(128) tc_scale_kernel(int D, int K, const float
         if (d < D && acc > 0.0 && isfinite(acc)) {
             const double e = rint(0.5 * log2(acc));
             s = (float)exp2(-fmin(fmax(e, -60.0), 60.0));
-            kp = (float)(accm * (double)s * (double)s);      // mean of mu^2 in scaled units
+            kp = (float)(accm * (double)s * (double)s);      // mean of (mu - g)^2 in scaled units
         }
         sd[d] = s;
         kap[d] = kp;
+        gd[d] = (float)g;
     }
 }
 
@@ -1188,7 +1233,7 @@ __global__ void __launch_bounds__(128) tc_scale_kernel(int D, int K, const float
 __global__ void __launch_bounds__(128) tc_prepare_kernel(int D, int K, const float* __restrict__ pi,
                                                          const float* __restrict__ mu, const float* __restrict__ var,
                                                          const float* __restrict__ sd, const float* __restrict__ kap,
-                                                         uint32_t* __restrict__ phi_img,
+                                                         const float* __restrict__ gd, uint32_t* __restrict__ phi_img,
                                                          unsigned char* __restrict__ plo_img, float* __restrict__ tk,
                                                          float* __restrict__ ck, float* __restrict__ illb, float cond_limit,
                                                          int* __restrict__ flags, uint32_t* __restrict__ phi_rm,
@@ -1200,7 +1245,7 @@ __global__ void __launch_bounds__(128) tc_prepare_kernel(int D, int K, const flo
     double a = 0.0, b = 0.0, cterm = 0.0, cond = 0.0;
     const bool live = (k < K) && (d < D);
     if (live) {
-        const double v = (double)var[(size_t)k * D + d], m = (double)mu[(size_t)k * D + d], s = (double)sd[d];
+        const double v = (double)var[(size_t)k * D + d], m = (double)mu[(size_t)k * D + d] - (double)gd[d], s = (double)sd[d];
         const double w = 1.4426950408889634074 / v;
         a = w * m / s;
         b = -0.5 * w / (s * s);
@@ -1278,11 +1323,11 @@ __global__ void __launch_bounds__(128) tc_prepare_kernel(int D, int K, const flo
 }
 
 // One warp per ill-conditioned component (illb > 0): its 8 dimensions of largest weight, in descending order of the weight,
-// in units of the scaled data (the tile kernel reads s_d x from the fp16 planes): weight (log2 e / 2) / (var s_d^2), mean
-// s_d mu.  The tile kernel uses them for an exact upper bound of log2 z that costs a few shared-memory reads.
+// in units of the centred, scaled data (the tile kernel reads s_d (x - g_d) from the fp16 planes): weight
+// (log2 e / 2) / (var s_d^2), mean s_d (mu - g_d).  The tile kernel uses them for an exact upper bound of log2 z that costs a few shared-memory reads.
 __global__ void __launch_bounds__(256) tc_decisive_kernel(int D, int K, const float* __restrict__ mu, const float* __restrict__ var,
-                                                          const float* __restrict__ sd, const float* __restrict__ illb,
-                                                          int* __restrict__ dec_dim, float* __restrict__ dec_w,
+                                                          const float* __restrict__ sd, const float* __restrict__ gd,
+                                                          const float* __restrict__ illb, int* __restrict__ dec_dim, float* __restrict__ dec_w,
                                                           float* __restrict__ dec_mu) {
     const int k = (int)((blockIdx.x * blockDim.x + threadIdx.x) >> 5), lane = threadIdx.x & 31;
     if (k >= K || !(illb[k] > 0.f)) return;          // warp-uniform
@@ -1318,7 +1363,7 @@ __global__ void __launch_bounds__(256) tc_decisive_kernel(int D, int K, const fl
             const bool have = bv >= 0.f;
             dec_dim[k * 8 + r] = have ? bd : 0;
             dec_w[k * 8 + r] = have ? bv : 0.f;
-            dec_mu[k * 8 + r] = have ? sd[bd] * mu[(size_t)k * D + bd] : 0.f;
+            dec_mu[k * 8 + r] = have ? sd[bd] * (mu[(size_t)k * D + bd] - gd[bd]) : 0.f;
         }
     }
 }
@@ -1386,37 +1431,44 @@ __global__ void __launch_bounds__(TC_MAX_ILL) tc_ill_cache_kernel(int D, const f
 }
 
 // stats (+)= sum over Q cluster partials (float64, fixed order), undoing the responsibility scale, the per-dimension
-// data scale and the interleaved column order.
+// data scale and centre, and the interleaved column order.
 __global__ void tc_reduce_kernel(int D, int K, int Kpad, int Q, const double* __restrict__ partial,
-                                 const float* __restrict__ sd, const float* __restrict__ kap, double* __restrict__ Nk,
-                                 double* __restrict__ S1, double* __restrict__ S2, int accumulate) {
+                                 const float* __restrict__ sd, const float* __restrict__ kap, const float* __restrict__ gd,
+                                 double* __restrict__ Nk, double* __restrict__ S1, double* __restrict__ S2, int accumulate) {
     const size_t KD = (size_t)K * D, per = (size_t)K + 2 * KD;
     const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (e >= per) return;
-    int k, col;
-    double unscale = 1.0 / (double)TC_RSCALE;
-    double* dst;
+    const double unscale = 1.0 / (double)TC_RSCALE;
+    auto column = [&](int col, int k) {                      // fixed order over the CTA groups
+        double s = 0.0;
+        for (int q = 0; q < Q; ++q) s += partial[((size_t)q * TC_PCOLS + col) * Kpad + k];
+        return s;
+    };
     if (e < (size_t)K) {
-        k = (int)e; col = 256; dst = Nk + e;     // plus column 257 (second softmax group), added below
-    } else if (e < K + KD) {
-        const size_t j = e - K; k = (int)(j / D); const int d = (int)(j % D);
-        col = 16 * (d >> 3) + (d & 7); unscale /= (double)sd[d]; dst = S1 + j;
+        const int k = (int)e;
+        const double s = (column(256, k) + column(257, k)) * unscale;      // N_k of the two softmax groups
+        Nk[e] = accumulate ? (Nk[e] + s) : s;
+        return;
+    }
+    // The planes hold u = s_d (x - g_d) and u^2 + kap_d: the sums come back as S1c = sum r (x - g), S2c = sum r (x - g)^2,
+    // then  S1 = S1c + g N_k,  S2 = S2c + 2 g S1c + g^2 N_k.
+    const bool second = e >= K + KD;
+    const size_t j = second ? (e - K - KD) : (e - K);
+    const int k = (int)(j / D), d = (int)(j % D);
+    const int col = 16 * (d >> 3) + (d & 7);
+    const double s_d = (double)sd[d], g = (double)gd[d];
+    const double nk_raw = column(256, k) + column(257, k);
+    const double nk = nk_raw * unscale;
+    const double s1c = column(col, k) * unscale / s_d;
+    double out;
+    if (!second) {
+        out = s1c + g * nk;
     } else {
-        const size_t j = e - K - KD; k = (int)(j / D); const int d = (int)(j % D);
-        col = 16 * (d >> 3) + (d & 7) + 8; unscale /= (double)sd[d] * (double)sd[d]; dst = S2 + j;
+        const double s2c = (column(col + 8, k) - (double)kap[d] * nk_raw) * unscale / (s_d * s_d);
+        out = s2c + 2.0 * g * s1c + g * g * nk;
     }
-    double s = 0.0;
-    for (int q = 0; q < Q; ++q) s += partial[((size_t)q * TC_PCOLS + col) * Kpad + k];
-    if (e < (size_t)K)
-        for (int q = 0; q < Q; ++q) s += partial[((size_t)q * TC_PCOLS + 257) * Kpad + k];
-    if (e >= K + KD) {          // squares were accumulated as (s x)^2 + kap: take kap * N_k out again
-        const int d = (int)((e - K - KD) % D);
-        double nk = 0.0;
-        for (int q = 0; q < Q; ++q) nk += partial[((size_t)q * TC_PCOLS + 256) * Kpad + k] + partial[((size_t)q * TC_PCOLS + 257) * Kpad + k];
-        s -= (double)kap[d] * nk;
-    }
-    s *= unscale;
-    *dst = accumulate ? (*dst + s) : s;
+    double* dst = second ? (S2 + j) : (S1 + j);
+    *dst = accumulate ? (*dst + out) : out;
 }
 
 // Fisher vectors of the groups of a grouped launch, straight from the per-CTA-group partials (group b of the launch =
@@ -1425,6 +1477,7 @@ __global__ void tc_reduce_kernel(int D, int K, int Kpad, int Q, const double* __
 // in float64.  out_index[b] = which of the caller's groups it is, group_points[b] = its T.
 __global__ void __launch_bounds__(256) tc_fisher_kernel(int D, int K, int Kpad, const double* __restrict__ partial,
                                                         const float* __restrict__ sd, const float* __restrict__ kap,
+                                                        const float* __restrict__ gd,
                                                         const float* __restrict__ pi, const float* __restrict__ mu,
                                                         const float* __restrict__ var, const int* __restrict__ out_index,
                                                         const int64_t* __restrict__ group_points, float* __restrict__ fv) {
@@ -1467,7 +1520,8 @@ __global__ void __launch_bounds__(256) tc_fisher_kernel(int D, int K, int Kpad, 
         float gm = 0.f, gs = 0.f;
         if (w > 0.f) {
             const float vf = var[e];
-            const double m = (double)mu[e], v = (double)vf;
+            // s1, s2 are moments of x - g: the vector depends on x - mu only, so the centred mean is used with them
+            const double m = (double)mu[e] - (double)gd[d], v = (double)vf;
             gm = (float)(s1 - m * nk) * (inv_t * rsqrtf(vf) * rsqrtf(w));
             gs = (float)((s2 - 2.0 * m * s1) + (m * m - v) * nk) * (inv_t * rsqrtf(2.0f * w) / vf);
         }
@@ -1482,16 +1536,16 @@ cudaError_t launch_fisher_tc(cudaStream_t s, int D, int K, int groups, const TcB
                              const float* var, const int* out_index, const int64_t* group_points, float* fv) {
     const TcPlan pl = tc_plan(D, K, 148);
     tc_fisher_kernel<<<dim3((unsigned)((K + 31) / 32), (unsigned)((D + 31) / 32), (unsigned)groups), 256, 0, s>>>(
-        D, K, pl.Kpad, tb.partial, tb.sd, tb.kap, pi, mu, var, out_index, group_points, fv);
+        D, K, pl.Kpad, tb.partial, tb.sd, tb.kap, tb.gd, pi, mu, var, out_index, group_points, fv);
     return cudaGetLastError();
 }
 
 cudaError_t launch_transform_grouped_tc(cudaStream_t s, const float* X, int64_t rows, int D, const int* tile_valid,
-                                        const int64_t* tile_src, const TcBuffers& tb) {
+                                        const int64_t* tile_src, const TcBuffers& tb, int* status) {
     if (rows < 1 || rows > TC_YPOINTS || rows % TC_BN != 0) return cudaErrorInvalidValue;
     int64_t blocks = (rows * 16 + 255) / 256;
     if (blocks > 148 * 16) blocks = 148 * 16;
-    tc_transform_grouped_kernel<<<(unsigned)blocks, 256, 0, s>>>(X, rows, D, tile_valid, tile_src, tb.sd, tb.kap, tb.y_hi, tb.y_lo);
+    tc_transform_grouped_kernel<<<(unsigned)blocks, 256, 0, s>>>(X, rows, D, tile_valid, tile_src, tb.sd, tb.kap, tb.gd, tb.y_hi, tb.y_lo, status);
     return cudaGetLastError();
 }
 
@@ -1538,15 +1592,15 @@ cudaError_t launch_prepare_tc(cudaStream_t s, int D, int K, const float* pi, con
     (void)status;
     cudaError_t e0 = cudaMemsetAsync(tb.flags, 0, 8 * sizeof(int), s);
     if (e0 != cudaSuccess) return e0;
-    tc_scale_kernel<<<128, 128, 0, s>>>(D, K, pi, mu, var, tb.sd, tb.kap);
+    tc_scale_kernel<<<128, 128, 0, s>>>(D, K, pi, mu, var, tb.sd, tb.kap, tb.gd);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    tc_prepare_kernel<<<pl.Kpad, 128, 0, s>>>(D, K, pi, mu, var, tb.sd, tb.kap, tb.phi_img, tb.plo_img, tb.tk, tb.ck, tb.illb, cond_limit, tb.flags,
+    tc_prepare_kernel<<<pl.Kpad, 128, 0, s>>>(D, K, pi, mu, var, tb.sd, tb.kap, tb.gd, tb.phi_img, tb.plo_img, tb.tk, tb.ck, tb.illb, cond_limit, tb.flags,
                                                   reinterpret_cast<uint32_t*>(tb.p_hi_rm), reinterpret_cast<uint32_t*>(tb.p_lo_rm),
                                                   reinterpret_cast<float2*>(tb.tkck));
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    tc_decisive_kernel<<<(unsigned)((K + 7) / 8), 256, 0, s>>>(D, K, mu, var, tb.sd, tb.illb, tb.dec_dim, tb.dec_w, tb.dec_mu);
+    tc_decisive_kernel<<<(unsigned)((K + 7) / 8), 256, 0, s>>>(D, K, mu, var, tb.sd, tb.gd, tb.illb, tb.dec_dim, tb.dec_w, tb.dec_mu);
     e = cudaGetLastError();
     if (e != cudaSuccess || !ill_list) return e;
     tc_ill_list_kernel<<<1, 1024, 0, s>>>(pl.Kpad, tb.illb, tb.ill_list, tb.flags);
@@ -1558,13 +1612,13 @@ cudaError_t launch_ill_cache_tc(cudaStream_t s, int D, const float* mu, const fl
     return cudaGetLastError();
 }
 
-cudaError_t launch_transform_tc(cudaStream_t s, const float* X, int64_t n, int D, const TcBuffers& tb) {
+cudaError_t launch_transform_tc(cudaStream_t s, const float* X, int64_t n, int D, const TcBuffers& tb, int* status) {
     if (n < 1 || n > TC_YPOINTS) return cudaErrorInvalidValue;
     const int64_t rows_padded = (n + TC_BN - 1) / TC_BN * TC_BN;
     const int64_t units = rows_padded * 16;
     int64_t blocks = (units + 255) / 256;
     if (blocks > 148 * 16) blocks = 148 * 16;
-    tc_transform_kernel<<<(unsigned)blocks, 256, 0, s>>>(X, n, rows_padded, D, tb.sd, tb.kap, tb.y_hi, tb.y_lo);
+    tc_transform_kernel<<<(unsigned)blocks, 256, 0, s>>>(X, n, rows_padded, D, tb.sd, tb.kap, tb.gd, tb.y_hi, tb.y_lo, status);
     return cudaGetLastError();
 }
 
@@ -1687,7 +1741,7 @@ cudaError_t launch_reduce_tc(cudaStream_t s, int D, int K, int Q, const TcBuffer
                              double* S2, bool accumulate) {
     const TcPlan pl = tc_plan(D, K, 148);
     const size_t per = (size_t)K + 2 * (size_t)K * D;
-    tc_reduce_kernel<<<(unsigned)((per + 255) / 256), 256, 0, s>>>(D, K, pl.Kpad, Q, tb.partial, tb.sd, tb.kap, Nk, S1, S2, accumulate ? 1 : 0);
+    tc_reduce_kernel<<<(unsigned)((per + 255) / 256), 256, 0, s>>>(D, K, pl.Kpad, Q, tb.partial, tb.sd, tb.kap, tb.gd, Nk, S1, S2, accumulate ? 1 : 0);
     return cudaGetLastError();
 }
 

@@ -39,6 +39,7 @@ struct TcBuffers {
     float* ck;
     float* sd;
     float* kap;
+    float* gd;      // [128] per-dimension centre subtracted from points and means (0 for padded dimensions)
     float* illb;
     int* flags;
     double* partial;
@@ -68,7 +69,8 @@ cudaError_t tc_max_clusters(int D, int K, int* out);
 cudaError_t launch_prepare_tc(cudaStream_t s, int D, int K, const float* pi, const float* mu, const float* var,
                               const TcBuffers& tb, float cond_limit, int* status, bool ill_list = false);
 // One pass over at most TC_YPOINTS points: X -> the two fp16 planes of Y in scratch (read by the tile kernel through TMA).
-cudaError_t launch_transform_tc(cudaStream_t s, const float* X, int64_t n, int D, const TcBuffers& tb);
+// A non-finite value in X raises ST_BAD_X in *status (the planes themselves are clamped to a finite range).
+cudaError_t launch_transform_tc(cudaStream_t s, const float* X, int64_t n, int D, const TcBuffers& tb, int* status);
 // n <= TC_YPOINTS points whose planes launch_transform_tc has written.
 // mu, w2, c2: the FP32 path's derived parameters (launch_prepare_fp32), used to recompute ill-conditioned logits exactly.
 // tight: use the filter meant for launches in which many components are ill-conditioned (tb.flags[4] counts them).
@@ -80,7 +82,7 @@ cudaError_t launch_em_tc(cudaStream_t s, const float* X, int64_t n, int D, int K
 // group's statistics in partial[b].  tile_valid[t] (0 .. TC_BN) = points of tile t, tile_src[t] = their first row in X
 // (device arrays, rows / TC_BN entries); launch_em_tc then gets n = rows and the same two arrays.
 cudaError_t launch_transform_grouped_tc(cudaStream_t s, const float* X, int64_t rows, int D, const int* tile_valid,
-                                        const int64_t* tile_src, const TcBuffers& tb);
+                                        const int64_t* tile_src, const TcBuffers& tb, int* status);
 // After a grouped launch_em_tc: Fisher vector of group b (its T = group_points[b]) into fv[out_index[b]][2][K][D].
 cudaError_t launch_fisher_tc(cudaStream_t s, int D, int K, int groups, const TcBuffers& tb, const float* pi, const float* mu,
                              const float* var, const int* out_index, const int64_t* group_points, float* fv);

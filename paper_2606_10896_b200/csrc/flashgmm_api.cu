@@ -18,8 +18,9 @@ namespace {
 
 struct DevResult {
     double ll[LL_SLOTS];
-    int status;
+    int status;     // sticky: device code ORs bits in; the host clears it only after it has reported them
     int n_ill;      // ill-conditioned components found by the tensor path's last preparation
+    int counts[2];  // the last parameter update: variance entries raised to the floor, components left unchanged as empty
 };
 
 constexpr size_t STAGE_BYTES = (size_t)128 << 20;   // per staging buffer of the host-streaming path
@@ -29,7 +30,7 @@ inline size_t align256(size_t b) { return (b + 255) & ~(size_t)255; }
 
 struct ScratchLayout {
     size_t w2, c2, c2d, center, partials, logZ2, llpart, result, stats, total;
-    size_t tc_phi, tc_plo, tc_tk, tc_ck, tc_sd, tc_kap, tc_illb, tc_flags, tc_xg, tc_xl, tc_partial, tc_llpart, tc_partial_bytes, tc_yhi, tc_ylo, tc_phirm, tc_plorm, tc_tkck, tc_illlist, tc_illcache, tc_decdim, tc_decw, tc_decmu;
+    size_t tc_phi, tc_plo, tc_tk, tc_ck, tc_sd, tc_kap, tc_gd, tc_illb, tc_flags, tc_xg, tc_xl, tc_partial, tc_llpart, tc_partial_bytes, tc_yhi, tc_ylo, tc_phirm, tc_plorm, tc_tkck, tc_illlist, tc_illcache, tc_decdim, tc_decw, tc_decmu;
     bool tc;
 };
 
@@ -49,7 +50,7 @@ ScratchLayout scratch_layout(int D, int K, bool planes) {
     L.result = take(sizeof(DevResult));
     L.stats = take(((size_t)K + 2 * KD) * 8);
     L.tc = tc_assign_supports(D, K);           // the assignment kernels' shapes include the E+M tile kernel's
-    L.tc_phi = L.tc_plo = L.tc_tk = L.tc_ck = L.tc_sd = L.tc_kap = L.tc_illb = L.tc_flags = L.tc_xg = L.tc_xl = L.tc_partial = L.tc_llpart = L.tc_yhi = L.tc_ylo = L.tc_phirm = L.tc_plorm = L.tc_tkck = L.tc_illlist = L.tc_illcache = L.tc_decdim = L.tc_decw = L.tc_decmu = 0;
+    L.tc_phi = L.tc_plo = L.tc_tk = L.tc_ck = L.tc_sd = L.tc_kap = L.tc_gd = L.tc_illb = L.tc_flags = L.tc_xg = L.tc_xl = L.tc_partial = L.tc_llpart = L.tc_yhi = L.tc_ylo = L.tc_phirm = L.tc_plorm = L.tc_tkck = L.tc_illlist = L.tc_illcache = L.tc_decdim = L.tc_decw = L.tc_decmu = 0;
     L.tc_partial_bytes = 0;
     if (L.tc) {
         const TcPlan pl = tc_plan(D, K, 160);       // an upper bound on the number of clusters
@@ -59,6 +60,7 @@ ScratchLayout scratch_layout(int D, int K, bool planes) {
         L.tc_ck = take((size_t)pl.Kpad * 4);
         L.tc_sd = take(128 * 4);
         L.tc_kap = take(128 * 4);
+        L.tc_gd = take(128 * 4);
         L.tc_illb = take((size_t)pl.Kpad * 4);
         L.tc_flags = take(32);
         if (tc_supports(D, K)) {                // what only the E+M tile kernel needs
@@ -116,6 +118,7 @@ struct gmm_ctx {
     int64_t tc_piece = TC_YPOINTS;   // points per launch of the tile kernel (<= capacity of the Y planes)
     int tc_n_ill = 0;                // ill-conditioned components at the last result that was read back (picks the filter)
     int tc_force_filter = -1;        // GMM_TC_FILTER=plain / tight: 0 / 1 (tests); -1: automatic
+    int sticky_status = 0;           // status bits read off the device but not yet reported (see ensure_scratch)
     // host-streaming path
     cudaStream_t copy_stream = nullptr;
     float* xstage[2] = {nullptr, nullptr};
@@ -149,6 +152,7 @@ struct gmm_ctx {
         b.ck = reinterpret_cast<float*>(scratch + lay.tc_ck);
         b.sd = reinterpret_cast<float*>(scratch + lay.tc_sd);
         b.kap = reinterpret_cast<float*>(scratch + lay.tc_kap);
+        b.gd = reinterpret_cast<float*>(scratch + lay.tc_gd);
         b.illb = reinterpret_cast<float*>(scratch + lay.tc_illb);
         b.flags = reinterpret_cast<int*>(scratch + lay.tc_flags);
         b.xg = scratch + lay.tc_xg;
@@ -205,9 +209,15 @@ int ensure_scratch(gmm_ctx* ctx, int D, int K) {
     const bool planes = tc_assign_supports(D, K) && (ctx->path == GMM_PATH_TENSOR || (ctx->path == GMM_PATH_AUTO && auto_wants_planes(D, K)));
     if (ctx->scratch && D == ctx->capD && K == ctx->capK && planes == ctx->capPlanes) return GMM_OK;
     const ScratchLayout L = scratch_layout(D, K, planes);
+    if (ctx->scratch) {
+        // The status word moves with the layout: what asynchronous calls may have left in it is kept on the host.
+        int st = 0;
+        CU(cudaMemcpyAsync(&st, &ctx->result()->status, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
+        CU(cudaStreamSynchronize(ctx->stream));
+        ctx->sticky_status |= st;
+    }
     if (L.total > ctx->scratch_bytes) {
         if (ctx->scratch) {
-            CU(cudaStreamSynchronize(ctx->stream));
             CU(cudaFree(ctx->scratch));
             ctx->scratch = nullptr;
             ctx->scratch_bytes = 0;
@@ -225,6 +235,7 @@ int ensure_scratch(gmm_ctx* ctx, int D, int K) {
     ctx->capD = D;
     ctx->capK = K;
     ctx->capPlanes = planes;
+    CU(cudaMemsetAsync(ctx->result(), 0, sizeof(DevResult), ctx->stream));
     ctx->tc_Q = 0;
     if (L.tc && tc_supports(D, K)) {
         int q = 0;
@@ -289,7 +300,6 @@ int prof_end(gmm_ctx* ctx) {
 // path: the tensor-core path whenever the shape allows it (ill-conditioned components are handled inside its kernel).
 int prepare_and_choose(gmm_ctx* ctx, int64_t N, int D, int K, const float* pi, const float* mu, const float* var,
                        int* path) {
-    CU(cudaMemsetAsync(&ctx->result()->status, 0, sizeof(int), ctx->stream));
     KL(launch_prepare_fp32(ctx->stream, D, K, pi, mu, var, ctx->w2(), ctx->c2(), ctx->c2d(), ctx->center(), &ctx->result()->status));
     if ((size_t)K * D > ((size_t)1 << 12)) ctx->launches++;      // but for tiny problems, the centre of the means is a launch of its own
     const bool tc_ok = ctx->lay.tc && ctx->tc_Q >= 1;
@@ -339,7 +349,7 @@ int accumulate_points(gmm_ctx* ctx, int path, const float* X, int64_t n, int D, 
             const int64_t cnt = (n - off < ctx->tc_piece) ? (n - off) : ctx->tc_piece;
             const float* Xs = X + off * D;
             CHECK(prof_begin(ctx));
-            KL(launch_transform_tc(ctx->stream, Xs, cnt, D, tb));
+            KL(launch_transform_tc(ctx->stream, Xs, cnt, D, tb, &ctx->result()->status));
             KL(launch_em_tc(ctx->stream, Xs, cnt, D, K, mu, ctx->w2(), ctx->c2(), tb, Q, ctx->tc_flush, tight, &ctx->result()->status));
             CHECK(prof_end(ctx));
         }
@@ -356,7 +366,7 @@ int accumulate_points(gmm_ctx* ctx, int path, const float* X, int64_t n, int D, 
         KL(launch_mstep_fp32(ctx->stream, Xs, cnt, D, K, mu, ctx->w2(), ctx->c2d(), ctx->center(), ctx->logZ2(), ctx->partials(), plan));
         CHECK(prof_end(ctx));
         KL(launch_reduce_ll(ctx->stream, ctx->llpart(), (cnt + FP32_TILE_P - 1) / FP32_TILE_P, &ctx->result()->ll[slot], true));
-        KL(launch_reduce_partials(ctx->stream, D, K, plan.splits, ctx->partials(), Nk, S1, S2, true));
+        KL(launch_reduce_partials(ctx->stream, D, K, plan.splits, ctx->partials(), ctx->center(), Nk, S1, S2, true));
     }
     return GMM_OK;
 }
@@ -370,18 +380,30 @@ int zero_stats(gmm_ctx* ctx, int D, int K, double* Nk, double* S1, double* S2, i
     return GMM_OK;
 }
 
+// The status word is sticky: device code ORs error bits into it and nothing clears it until the host has reported
+// them, so an error raised by an asynchronous call (gmm_assign_topm, gmm_finalize) surfaces at the next synchronising
+// call or at gmm_sync_status.  Called with the stream synchronised and `status` = the word as read from the device.
+int report_status(gmm_ctx* ctx, int status) {
+    status |= ctx->sticky_status;
+    if (status == 0) return GMM_OK;
+    ctx->sticky_status = 0;
+    CU(cudaMemsetAsync(&ctx->result()->status, 0, sizeof(int), ctx->stream));
+    if (status & ST_TIMEOUT) return fail(ctx, GMM_ETIMEOUT, "a bounded device-side wait expired (in this call or an earlier asynchronous one)");
+    if (status & ST_BAD_VAR) return fail(ctx, GMM_ENUMERIC, "var must be finite and > 0 (in this call or an earlier asynchronous one)");
+    if (status & ST_BAD_PI) return fail(ctx, GMM_ENUMERIC, "pi must be finite and >= 0 (in this call or an earlier asynchronous one)");
+    if (status & ST_BAD_X) return fail(ctx, GMM_ENUMERIC, "X holds a non-finite value (in this call or an earlier asynchronous one)");
+    return fail(ctx, GMM_ENUMERIC, "non-finite parameter (in this call or an earlier asynchronous one)");
+}
+
 // Synchronising read of the log-likelihood slot and the status word.
 int read_result(gmm_ctx* ctx, int slot, double* loglik) {
     DevResult r;
     CU(cudaMemcpyAsync(&r, ctx->result(), sizeof(DevResult), cudaMemcpyDeviceToHost, ctx->stream));
     CU(cudaStreamSynchronize(ctx->stream));
-    if (r.status & ST_TIMEOUT) return fail(ctx, GMM_ETIMEOUT, "a bounded device-side wait expired");
-    if (r.status & ST_BAD_VAR) return fail(ctx, GMM_ENUMERIC, "var must be finite and > 0");
-    if (r.status & ST_BAD_PI) return fail(ctx, GMM_ENUMERIC, "pi must be finite and >= 0");
-    if (r.status & ST_NONFINITE) return fail(ctx, GMM_ENUMERIC, "non-finite parameter");
+    CHECK(report_status(ctx, r.status));
     ctx->tc_n_ill = r.n_ill;
     *loglik = r.ll[slot];
-    if (!std::isfinite(*loglik)) return fail(ctx, GMM_ENUMERIC, "log-likelihood is not finite (%g)", *loglik);
+    if (!std::isfinite(*loglik)) return fail(ctx, GMM_ENUMERIC, "log-likelihood is not finite (%g): non-finite values in X?", *loglik);
     return GMM_OK;
 }
 
@@ -502,7 +524,9 @@ int gmm_finalize(gmm_ctx* ctx, int64_t N, int D, int K, const double* Nk, const 
     CHECK(check_ptr(ctx, var, 4, "var"));
     if (!(var_floor >= 0.f)) return fail(ctx, GMM_EINVAL, "var_floor must be >= 0");
     DeviceGuard g(ctx->device);
-    KL(launch_finalize(ctx->stream, N, D, K, Nk, S1, S2, var_floor, pi, mu, var));
+    int* counts = ctx->scratch ? ctx->result()->counts : nullptr;
+    if (counts) CU(cudaMemsetAsync(counts, 0, 2 * sizeof(int), ctx->stream));
+    KL(launch_finalize(ctx->stream, N, D, K, Nk, S1, S2, var_floor, pi, mu, var, counts, nullptr, nullptr));
     return GMM_OK;
 }
 
@@ -524,7 +548,9 @@ int gmm_finalize_isotropic(gmm_ctx* ctx, int64_t N, int D, int K, const double* 
     CHECK(check_ptr(ctx, var, 4, "var"));
     if (!(var_floor >= 0.f)) return fail(ctx, GMM_EINVAL, "var_floor must be >= 0");
     DeviceGuard g(ctx->device);
-    KL(launch_finalize_isotropic(ctx->stream, N, D, K, Nk, S1, S2, var_floor, pi, mu, var));
+    int* counts = ctx->scratch ? ctx->result()->counts : nullptr;
+    if (counts) CU(cudaMemsetAsync(counts, 0, 2 * sizeof(int), ctx->stream));
+    KL(launch_finalize_isotropic(ctx->stream, N, D, K, Nk, S1, S2, var_floor, pi, mu, var, counts, nullptr, nullptr));
     return GMM_OK;
 }
 
@@ -552,10 +578,15 @@ int gmm_fit(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, float* pi, fl
         CHECK(prepare_and_choose(ctx, N, D, K, pi, mu, var, &path));
         CHECK(zero_stats(ctx, D, K, Nk, S1, S2, slot));
         CHECK(accumulate_points(ctx, path, X, N, D, K, mu, Nk, S1, S2, slot));
+        // The update is skipped on the device when the step raised a status bit or left a non-finite log-likelihood
+        // (invalid parameters, a time-out, non-finite data): the caller then keeps the last good parameters.
+        CU(cudaMemsetAsync(ctx->result()->counts, 0, 2 * sizeof(int), ctx->stream));
         if (ctx->covariance == GMM_COV_ISOTROPIC)
-            KL(launch_finalize_isotropic(ctx->stream, N, D, K, Nk, S1, S2, var_floor, pi, mu, var));
+            KL(launch_finalize_isotropic(ctx->stream, N, D, K, Nk, S1, S2, var_floor, pi, mu, var, ctx->result()->counts,
+                                         &ctx->result()->status, &ctx->result()->ll[slot]));
         else
-            KL(launch_finalize(ctx->stream, N, D, K, Nk, S1, S2, var_floor, pi, mu, var));
+            KL(launch_finalize(ctx->stream, N, D, K, Nk, S1, S2, var_floor, pi, mu, var, ctx->result()->counts,
+                               &ctx->result()->status, &ctx->result()->ll[slot]));
         ctx->last_path = path;
         int rc = read_result(ctx, slot, &loglik_trace[t]);
         if (rc != GMM_OK) {
@@ -676,7 +707,6 @@ namespace {
 // The assignment pass proper (arguments checked, scratch in place); also the nearest-centroid search of the k-means step.
 int assign_topm_impl(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const float* pi, const float* mu,
                      const float* var, int m, int32_t* idx, float* resp, bool index_only) {
-    CU(cudaMemsetAsync(&ctx->result()->status, 0, sizeof(int), ctx->stream));
     KL(launch_prepare_fp32(ctx->stream, D, K, pi, mu, var, ctx->w2(), ctx->c2(), ctx->c2d(), ctx->center(), &ctx->result()->status));
     if ((size_t)K * D > ((size_t)1 << 12)) ctx->launches++;      // but for tiny problems, the centre of the means is a launch of its own
     // Tensor-core assignment where the E+M step would take the tensor path too.  Ill-conditioned components are evaluated
@@ -710,7 +740,7 @@ int assign_topm_impl(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, cons
                 CU(cudaMemsetAsync(unc_count, 0, sizeof(int), ctx->stream));
             }
             CHECK(prof_begin(ctx));
-            KL(launch_transform_tc(ctx->stream, X + off * D, cnt, D, tb));
+            KL(launch_transform_tc(ctx->stream, X + off * D, cnt, D, tb, &ctx->result()->status));
             KL(launch_assign_tc(ctx->stream, X + off * D, cnt, D, K, mu, ctx->w2(), ctx->c2(), tb, reinterpret_cast<float*>(base),
                                 unc_rows, unc_count, (int)(off - win_start), m, idx + off * m, resp ? resp + off * m : nullptr, &ctx->result()->status,
                                 index_only));
@@ -879,7 +909,6 @@ int gmm_score_samples(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, con
     CHECK(check_ptr(ctx, logp, 4, "logp"));
     DeviceGuard guard(ctx->device);
     CHECK(ensure_scratch(ctx, D, K));
-    CU(cudaMemsetAsync(&ctx->result()->status, 0, sizeof(int), ctx->stream));
     KL(launch_prepare_fp32(ctx->stream, D, K, pi, mu, var, ctx->w2(), ctx->c2(), ctx->c2d(), ctx->center(), &ctx->result()->status));
     if ((size_t)K * D > ((size_t)1 << 12)) ctx->launches++;
     CU(cudaMemsetAsync(&ctx->result()->ll[0], 0, 8, ctx->stream));
@@ -1011,7 +1040,7 @@ int gmm_fisher_vectors(gmm_ctx* ctx, const float* X, int64_t N, const int64_t* o
                 CU(cudaMemsetAsync(tb.partial, 0, (size_t)bt.Q * pl.Kpad * TC_PCOLS * 8, ctx->stream));
                 CU(cudaMemsetAsync(tb.llpart, 0, (size_t)bt.Q * 16, ctx->stream));
                 CHECK(prof_begin(ctx));
-                KL(launch_transform_grouped_tc(ctx->stream, X, rows, D, d_valid + bt.tile0, d_src + bt.tile0, tb));
+                KL(launch_transform_grouped_tc(ctx->stream, X, rows, D, d_valid + bt.tile0, d_src + bt.tile0, tb, &ctx->result()->status));
                 KL(launch_em_tc(ctx->stream, X, rows, D, K, mu, ctx->w2(), ctx->c2(), tb, bt.Q, ctx->tc_flush, tight,
                                 &ctx->result()->status, d_valid + bt.tile0, d_src + bt.tile0));
                 CHECK(prof_end(ctx));
@@ -1039,15 +1068,39 @@ int gmm_fisher_vectors(gmm_ctx* ctx, const float* X, int64_t N, const int64_t* o
         DevResult r;
         CU(cudaMemcpyAsync(&r, ctx->result(), sizeof(DevResult), cudaMemcpyDeviceToHost, ctx->stream));
         CU(cudaStreamSynchronize(ctx->stream));
-        if (r.status & ST_BAD_VAR) return fail(ctx, GMM_ENUMERIC, "var must be finite and > 0");
-        if (r.status & ST_BAD_PI) return fail(ctx, GMM_ENUMERIC, "pi must be finite and >= 0");
-        if (r.status & ST_NONFINITE) return fail(ctx, GMM_ENUMERIC, "non-finite parameter");
+        CHECK(report_status(ctx, r.status));
         if (loglik) *loglik = 0.0;
         return GMM_OK;
     }
     const int rc = read_result(ctx, 0, &total);
     if (rc != GMM_OK) return rc;
     if (loglik) *loglik = total;
+    return GMM_OK;
+}
+
+int gmm_sync_status(gmm_ctx* ctx) {
+    if (!ctx) return GMM_EINVAL;
+    DeviceGuard g(ctx->device);
+    CU(cudaStreamSynchronize(ctx->stream));
+    int st = 0;
+    if (ctx->scratch) {
+        CU(cudaMemcpyAsync(&st, &ctx->result()->status, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
+        CU(cudaStreamSynchronize(ctx->stream));
+    }
+    if (st == 0 && ctx->sticky_status == 0) return GMM_OK;
+    return report_status(ctx, st);
+}
+
+int gmm_update_counts(gmm_ctx* ctx, int64_t* floored_variances, int64_t* empty_components) {
+    if (!ctx) return GMM_EINVAL;
+    DeviceGuard g(ctx->device);
+    int c[2] = {0, 0};
+    if (ctx->scratch) {
+        CU(cudaMemcpyAsync(c, ctx->result()->counts, sizeof(c), cudaMemcpyDeviceToHost, ctx->stream));
+        CU(cudaStreamSynchronize(ctx->stream));
+    }
+    if (floored_variances) *floored_variances = c[0];
+    if (empty_components) *empty_components = c[1];
     return GMM_OK;
 }
 

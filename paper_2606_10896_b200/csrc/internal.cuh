@@ -17,7 +17,7 @@ constexpr int FP32_TARGET_CTAS = 296;
 constexpr int LL_SLOTS = 64;       // device slots for log-likelihood values (gmm_fit keeps one per iteration in a ring)
 
 // Status word bits written by device code, read by the host after a synchronising call.
-enum : int { ST_BAD_VAR = 1, ST_BAD_PI = 2, ST_NONFINITE = 4, ST_TIMEOUT = 8, ST_ILLCOND = 16 };
+enum : int { ST_BAD_VAR = 1, ST_BAD_PI = 2, ST_NONFINITE = 4, ST_TIMEOUT = 8, ST_ILLCOND = 16, ST_BAD_X = 32 };
 
 struct Fp32Plan {
     int comp_blocks, d_chunks, splits;
@@ -51,16 +51,22 @@ cudaError_t launch_topm_fp32(cudaStream_t s, const float* X, int64_t n, int D, i
 
 // ---- shared by all paths -------------------------------------------------------------------------------------
 // stats (+)= sum over `splits` partial blocks, fixed order, float64.  Partial layout: [splits][K + 2*K*D] floats,
-// each block being (N_k [K], S1 [K*D], S2 [K*D]); float64 instead when fp32_plan(D, K).wide.
-cudaError_t launch_reduce_partials(cudaStream_t s, int D, int K, int splits, const float* partials, double* Nk,
-                                   double* S1, double* S2, bool accumulate);
+// each block being (N_k [K], sums of r (x - g) [K*D], sums of r (x - g)^2 [K*D]); float64 instead when
+// fp32_plan(D, K).wide.  g [D]: the centre launch_mstep_fp32 was given (NULL = 0); the shift back to S1, S2 is exact.
+cudaError_t launch_reduce_partials(cudaStream_t s, int D, int K, int splits, const float* partials, const float* g,
+                                   double* Nk, double* S1, double* S2, bool accumulate);
 // *ll (+)= sum of llpart[0..n) in a fixed order
 cudaError_t launch_reduce_ll(cudaStream_t s, const double* llpart, int64_t n, double* ll, bool accumulate);
+// counts (may be NULL): counts[0] += variance entries raised to the floor, counts[1] += components left unchanged
+// because N_k < 1e-12 (integer atomics).  skip_status / skip_ll (may be NULL): the kernel writes nothing when
+// *skip_status != 0 or *skip_ll is not finite (the step that produced the statistics failed).
 cudaError_t launch_finalize(cudaStream_t s, int64_t N, int D, int K, const double* Nk, const double* S1,
-                            const double* S2, float var_floor, float* pi, float* mu, float* var);
+                            const double* S2, float var_floor, float* pi, float* mu, float* var, int* counts,
+                            const int* skip_status, const double* skip_ll);
 
 cudaError_t launch_finalize_isotropic(cudaStream_t s, int64_t N, int D, int K, const double* Nk, const double* S1,
-                                      const double* S2, float var_floor, float* pi, float* mu, float* var);
+                                      const double* S2, float var_floor, float* pi, float* mu, float* var, int* counts,
+                                      const int* skip_status, const double* skip_ll);
 
 // ---- Fisher vector of one group from its statistics (paper Section 6) ----------------------------------------------
 // out[2 * K * D] (device): the means part [K x D], then the standard-deviations part [K x D]
@@ -75,7 +81,7 @@ size_t pl_scratch_bytes(int K);
 cudaError_t launch_posting_lists(cudaStream_t s, const int32_t* idx, const float* resp, int64_t n, int m, int K, float tau,
                                  int max_lists, void* scratch, int64_t* offsets, int32_t* items);
 
-// ---- one Lloyd (k-means) iteration: the paper's warm start (Section 5) -----------------------------------------------
+// ---- one Lloyd (k-means) iteration: the paper's warm start (Section 4.4 and the warm-start appendix) -----------------------------------------------
 size_t km_scratch_bytes(int D, int K);
 int64_t* km_offsets(void* scratch);                     // [K + 1] inside the scratch: the posting-list offsets go here
 double* km_inertia_k(void* scratch, int D, int K);      // [K] per-cluster inertia, written by launch_kmeans_update

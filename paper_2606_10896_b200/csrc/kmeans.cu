@@ -1,4 +1,4 @@
-// One Lloyd (k-means) iteration: the warm start the paper runs before its EM iterations (Section 5, experimental setup:
+// One Lloyd (k-means) iteration: the warm start the paper runs before its EM iterations (Section 4.4, experimental setup, and the warm-start appendix:
 // 10 iterations of k-means, then Flash-GMM).
 //
 // Assignment: the nearest centroid of a point is the top-1 "component" of a mixture with unit variances and equal

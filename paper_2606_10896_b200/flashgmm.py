@@ -67,6 +67,8 @@ EXPORTS = {
                                           ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                           ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                           ctypes.POINTER(ctypes.c_double)]),
+    "gmm_sync_status": (ctypes.c_int, [ctypes.c_void_p]),
+    "gmm_update_counts": (ctypes.c_int, [ctypes.c_void_p, ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int64)]),
     "gmm_scratch_bytes": (ctypes.c_size_t, [ctypes.c_int, ctypes.c_int]),
     "gmm_launch_count": (ctypes.c_int64, [ctypes.c_void_p]),
     "gmm_set_profiling": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int]),
@@ -204,6 +206,16 @@ class Context:
 
     def gmm_reset_counters(self):
         self._check(lib.gmm_reset_counters(self._h))
+
+    def gmm_sync_status(self):
+        """Waits for the stream; raises GmmError if an earlier asynchronous call recorded an error on the device."""
+        self._check(lib.gmm_sync_status(self._h))
+
+    def gmm_update_counts(self):
+        """(variance entries raised to the floor, components left unchanged as empty) of the last parameter update."""
+        fl, em = ctypes.c_int64(0), ctypes.c_int64(0)
+        self._check(lib.gmm_update_counts(self._h, ctypes.byref(fl), ctypes.byref(em)))
+        return int(fl.value), int(em.value)
 
     # ---- compute ----
     def gmm_em_step(self, X, pi, mu, var, out=None):

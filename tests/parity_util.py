@@ -32,15 +32,17 @@ def assert_params_close(N, s, got, ref, Nk_ref, what=""):
 
 def assert_stats_close(N, s, got, ref, what=""):
     """Statistics compared on the scale the parameter tolerances imply: N_k to 1e-5 N; S1 to 1e-4 s max(N_k, 1);
-    S2 to 1e-4 s^2 max(N_k, 1) plus the matching share of the mean term."""
+    S2 to 1e-4 s^2 max(N_k, 1) plus the matching share of the mean term.  The relative allowances are capped by the
+    data scale (10 s for a mean, 30 s^2 for a second moment), so that data far from the origin cannot widen them; what
+    decides is the parameter check after the update (assert_params_close)."""
     Nk_g, S1_g, S2_g = (np.asarray(a, np.float64) for a in got)
     Nk_r, S1_r, S2_r = ref
     assert np.abs(Nk_g - Nk_r).max() <= 1e-5 * N, f"{what}: N_k off by {np.abs(Nk_g - Nk_r).max():.3e}"
     w = np.maximum(Nk_r, 1.0)[:, None]
-    mean_abs = np.abs(S1_r) / w
+    mean_abs = np.minimum(np.abs(S1_r) / w, 10.0 * s)
     e1 = (np.abs(S1_g - S1_r) / w - 1e-5 * mean_abs).max()
     assert e1 <= 1e-4 * s, f"{what}: S1/N_k off by {e1:.3e} > {1e-4 * s:.3e}"
-    e2 = (np.abs(S2_g - S2_r) / w - 3e-5 * (S2_r / w)).max()
+    e2 = (np.abs(S2_g - S2_r) / w - 3e-5 * np.minimum(S2_r / w, 30.0 * s * s)).max()
     assert e2 <= 1e-4 * s * s, f"{what}: S2/N_k off by {e2:.3e} > {1e-4 * s * s:.3e}"
 
 

@@ -1,4 +1,4 @@
-"""One Lloyd (k-means) iteration, the paper's warm start (Section 5: 10 iterations of k-means before the EM iterations):
+"""One Lloyd (k-means) iteration, the paper's warm start (Section 4.4 and the warm-start appendix: 10 iterations of k-means before the EM iterations):
 pins of the CPU oracle, and parity of the CUDA step.
 
 The oracle (oracle/kmeans.py) is pinned by closed forms, by separated clusters whose answer is known by construction,

@@ -508,9 +508,10 @@ def test_topm_exact_ties_go_to_the_smaller_index(fg, ctx):
 
 
 def test_data_far_from_the_origin(fg, ctx):
-    """All points and means sit 300 standard deviations from the origin: the FP32 kernels form their products about the
-    centre of the means, so the offset costs no precision; the tensor path finds every component ill-conditioned for its
-    expanded form and recomputes what matters exactly."""
+    """All points and means sit 300 standard deviations from the origin.  Both paths form their products, and accumulate
+    their sums, about a per-dimension centre of the means and shift the statistics back in float64, so the offset costs
+    no precision: the updated parameters (whose variance is the cancelling difference S2 / N_k - mu^2, here 1 against
+    90,000) must meet the ordinary tolerances, and so must the raw statistics relative to their own size."""
     rng = np.random.default_rng(21)
     N, D, K = 4000, 64, 96
     X, pi, mu, var = _random_mixture(rng, N, D, K, spread=1.5)
@@ -518,14 +519,117 @@ def test_data_far_from_the_origin(fg, ctx):
     mu = (mu + 300.0).astype(np.float32)
     s = data_scale(X)
     ref = orc.em_step(X, pi, mu, var)
+    pr, mr, vr, _, _, _ = orc.em_iteration(X, pi, mu, var, var_floor=1e-6)
     for path in _paths(fg, D, K):
         ctx.gmm_set_path(path)
         got = _gpu_step(ctx, _t(X), pi, mu, var)
+        what = f"path {path}, data far from the origin"
         assert abs(got[3] - ref[3]) <= 1e-5 * abs(ref[3]), path
-        assert_stats_close(N, s, got[:3], ref[:3], f"path {path}, data far from the origin")
+        for g_, r_ in zip(got[:3], ref[:3]):            # raw statistics: 1e-6 of their own size
+            assert np.abs(g_ - r_).max() <= 1e-6 * np.abs(r_).max() + 1e-9, what
+        pi_d, mu_d, var_d = _t(pi), _t(mu), _t(var)
+        ctx.gmm_finalize(N, _t(got[0], torch.float64), _t(got[1], torch.float64), _t(got[2], torch.float64), 1e-6,
+                         pi_d, mu_d, var_d)
+        assert_params_close(N, s, (pi_d.cpu().numpy(), mu_d.cpu().numpy(), var_d.cpu().numpy()), (pr, mr, vr), ref[0], what)
         idx_g, resp_g = ctx.gmm_assign_topm(_t(X), _t(pi), _t(mu), _t(var), 3)
         torch.cuda.synchronize()
         _check_topm(X, pi, mu, var, 3, idx_g.cpu().numpy(), resp_g.cpu().numpy(), f"path {path}, far from the origin")
+
+
+def test_errors_of_asynchronous_calls_surface_at_the_next_synchronising_call(fg, ctx):
+    """gmm_assign_topm returns with its work in flight, so what its kernels find wrong (here var <= 0) cannot come back
+    as its return value: the device-side status word keeps it until gmm_sync_status, or the next call that synchronises,
+    reports it; the report clears it."""
+    rng = np.random.default_rng(5)
+    for D, K in ((16, 8), (64, 128)):                   # FP32 kernels; tensor-core assignment
+        X, pi, mu, var = _random_mixture(rng, 500, D, K)
+        bad = var.copy()
+        bad[K // 2, 3] = 0.0
+        with fg.Context(0) as c:
+            c.gmm_assign_topm(_t(X), _t(pi), _t(mu), _t(bad), 2)                # asynchronous: no error yet
+            with pytest.raises(fg.GmmError) as e:
+                c.gmm_sync_status()
+            assert e.value.code == fg.GMM_ENUMERIC
+            c.gmm_sync_status()                                                 # reported once, then clean
+            c.gmm_assign_topm(_t(X), _t(pi), _t(mu), _t(bad), 2)
+            with pytest.raises(fg.GmmError) as e:                               # ... or at the next synchronising call
+                c.gmm_em_step(_t(X), _t(pi), _t(mu), _t(var))
+            assert e.value.code == fg.GMM_ENUMERIC
+            Nk = c.gmm_em_step(_t(X), _t(pi), _t(mu), _t(var))[0]              # and the context stays usable
+            assert abs(float(Nk.sum()) - 500) < 1e-3
+
+
+def test_non_finite_data_is_reported_and_fit_keeps_the_last_good_parameters(fg, ctx):
+    rng = np.random.default_rng(6)
+    X, pi, mu, var = _random_mixture(rng, 3000, 32, 16)
+    for poison in (np.nan, np.inf):
+        Xb = X.copy()
+        Xb[1234, 5] = poison
+        for path in _paths(fg, 32, 16) + [fg.GMM_PATH_TENSOR]:
+            ctx.gmm_set_path(path)
+            with pytest.raises(fg.GmmError) as e:
+                ctx.gmm_em_step(_t(Xb), _t(pi), _t(mu), _t(var))
+            assert e.value.code == fg.GMM_ENUMERIC
+            pi_d, mu_d, var_d = _t(pi), _t(mu), _t(var)
+            with pytest.raises(fg.GmmError) as e:
+                ctx.gmm_fit(_t(Xb), pi_d, mu_d, var_d, 3)
+            assert e.value.code == fg.GMM_ENUMERIC
+            # the failed iteration's update was not applied
+            assert np.array_equal(mu_d.cpu().numpy(), mu) and np.array_equal(var_d.cpu().numpy(), var)
+            assert np.array_equal(pi_d.cpu().numpy(), pi)
+    ctx.gmm_set_path(fg.GMM_PATH_AUTO)
+    ctx.gmm_em_step(_t(X), _t(pi), _t(mu), _t(var))
+
+
+def test_fit_stops_on_the_relative_change_of_the_log_likelihood(fg, ctx):
+    """tol > 0 (the paper's "sufficiently small change", Section 2): the same stopping iteration as the oracle's loop."""
+    spec = synth.CONFIGS[1]
+    X = synth.sample_host(spec)
+    pi0, mu0, var0 = synth.init_params(X, spec)
+    tol = 2e-4
+    ref = orc.fit(X, pi0, mu0, var0, 40, var_floor=spec.var_floor)["trace"]
+    stop = next((t + 1 for t in range(1, len(ref)) if abs(ref[t] - ref[t - 1]) <= tol * abs(ref[t])), len(ref))
+    assert 2 <= stop < 40
+    for path in _paths(fg, spec.D, spec.K):
+        ctx.gmm_set_path(path)
+        trace, done = ctx.gmm_fit(_t(X), _t(pi0), _t(mu0), _t(var0), 40, spec.var_floor, tol=tol)
+        assert done == stop and len(trace) == stop
+        np.testing.assert_allclose(trace, ref[:stop], rtol=1e-4)
+
+
+def test_update_counts_report_floored_variances_and_empty_components(fg, ctx):
+    rng = np.random.default_rng(8)
+    N, D, K = 2000, 8, 5
+    X = rng.normal(size=(N, D)).astype(np.float32)
+    X[:, 0] = 2.0                                        # a constant dimension: every live component's variance there is 0
+    pi = np.array([0.5, 0.5, 0.0, 0.0, 0.0], np.float32)            # three components get no weight at all
+    mu = rng.normal(size=(K, D)).astype(np.float32)
+    var = np.ones((K, D), np.float32)
+    Nk, S1, S2, _ = ctx.gmm_em_step(_t(X), _t(pi), _t(mu), _t(var))
+    pi_d, mu_d, var_d = _t(pi), _t(mu), _t(var)
+    ctx.gmm_finalize(N, Nk, S1, S2, 1e-3, pi_d, mu_d, var_d)
+    assert ctx.gmm_update_counts() == (2, 3)
+    ctx.gmm_finalize_isotropic(N, Nk, S1, S2, 1e-3, pi_d, mu_d, var_d)
+    assert ctx.gmm_update_counts() == (0, 3)
+    pi_d, mu_d, var_d = _t(pi), _t(mu), _t(var)
+    ctx.gmm_fit(_t(X), pi_d, mu_d, var_d, 2, 1e-3)
+    assert ctx.gmm_update_counts() == (2, 3)
+
+
+def test_scratch_allocation_failure_is_reported_as_enomem(fg):
+    """All but 256 MB of the free device memory is taken before the first call that needs the 600 MB of scratch."""
+    free_b, _ = torch.cuda.mem_get_info()
+    hog = torch.empty(max(0, free_b - (256 << 20)), dtype=torch.uint8, device=DEV)
+    try:
+        X = _t(np.zeros((100, 128), np.float32))
+        K = 1024
+        with fg.Context(0) as c:
+            with pytest.raises(fg.GmmError) as e:
+                c.gmm_em_step(X, _t(np.full(K, 1 / K)), _t(np.zeros((K, 128))), _t(np.ones((K, 128))))
+            assert e.value.code == fg.GMM_ENOMEM
+    finally:
+        del hog
+        torch.cuda.empty_cache()
 
 
 @pytest.mark.parametrize("N,D,K", [(3000, 3, 1), (7001, 3, 5), (2000, 8, 2)])

@@ -1,0 +1,980 @@
+// Tensor-core path for wide data (128 < D <= 1024; sm_100a, tcgen05 + TMEM): the EM iteration in the two sweeps of the
+// paper's Algorithm 1, each a streamed contraction on the expanded quadratic form.
+//
+// Why two sweeps here and one for D <= 128: the M-step result of 128 components is 128 x 2D fp32 values, which for
+// D > 128 no longer fits the 512 TMEM columns of an SM next to the logits, and the coefficient slice of 128 components
+// (128 x 2D x 2 fp16 planes) no longer fits shared memory, so neither can stay on chip for the life of a CTA.
+//
+//   sweep 1  (lse_wide_kernel, TMEM lanes = POINTS)   Algorithm 1, Step 1.  A CTA takes tiles of 128 points and walks the
+//            components in groups of 512 (all 512 TMEM columns as accumulators); for every 64-column atom of the
+//            contraction it streams the tile's Y atom and the group's coefficient atoms through a ring in shared memory.
+//            A softmax thread owns one point: running (max, sum) over all K, log2 Z_i to a scratch buffer of one piece
+//            (2^17 points; no O(N) memory), sum of log2 Z for the log-likelihood.
+//   sweep 2  (em_wide_kernel, TMEM lanes = COMPONENTS)   Algorithm 1, Step 2.  A CTA owns 128 components and takes
+//            batches of 256 points: E-step again (main product and the two small cross products in separate TMEM
+//            accumulators), r = 2^(log2 z - log2 Z_i) written over the logits as fp16 hi + lo (the A operand of the
+//            M-step), then for each half-slice of 64 dimensions S[128 x 128] = r^T [Y | Y^2] over the batch in one of two
+//            alternating TMEM accumulators, which the softmax warps add to the CTA's own fp32 partial block in global
+//            memory while the next half-slice accumulates.  No exchange between CTAs and no cooperative launch: Z_i is
+//            known from sweep 1.
+// Precision as on the D <= 128 path (every operand split into two fp16 values; three products per contraction), with
+// kap_d chosen so that a component's own points give terms of zero mean in every dimension: the accumulators then stay
+// small (tens, not D / 2), and with them the truncation error of the tensor core's fp32 accumulation.
+// Ill-conditioned components (error estimate above the limit) are not handled here: the host sends such parameter
+// sets to the FP32 kernels.
+#include "internal.cuh"
+#include "em_tc.cuh"
+#include "em_wide.cuh"
+
+#include <cuda.h>
+#include <cuda_fp16.h>
+#include <math_constants.h>
+
+#define TC_WAIT_LIMIT_NS 2000000000ull
+#include "tc_prims.cuh"
+
+namespace fg {
+
+namespace {
+
+constexpr int WT_THREADS = 320;            // 8 softmax warps, producer warp, MMA warp
+constexpr int WT_PRODUCER = 8, WT_MMA = 9;
+constexpr int SLOT = 32768;                // ring slot: [hi 16 KB | lo 16 KB] or one 32 KB atom of 256 rows
+constexpr float RSCALE = TC_RSCALE;
+
+// ------------------------------------------------------------------------------------------------------------------
+// Sweep 1
+constexpr int L_SLOTS = 7;
+constexpr int L_BAR = L_SLOTS * SLOT;
+constexpr int L_MERGE = L_BAR + 256;                // 128 x 8 bytes: (max, sum) pairs of warpgroup 1, later the log-likelihood terms
+constexpr int L_SMEM = L_MERGE + 1024 + 1024;
+enum { LB_FULL = 0, LB_EMPTY = L_SLOTS, LB_LFULL = 2 * L_SLOTS, LB_LEMPTY, LB_FINAL, LB_COUNT };
+
+struct LseParams {
+    int64_t n;
+    int NC;              // chunks of 128 components
+    int NZ;              // atoms of 64 columns in the contraction (4 per slice of 128 dimensions)
+    const float2* tkck;  // [NC * 128]
+    const double* cref;
+    double* logz;
+    double* llpart;
+    int* status;
+};
+
+__global__ void __launch_bounds__(WT_THREADS, 1)
+lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, const __grid_constant__ CUtensorMap tm_ylo,
+                const __grid_constant__ CUtensorMap tm_phi, const __grid_constant__ CUtensorMap tm_plo) {
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int abort_s, drain_s;
+    volatile int* abort_flag = &abort_s;
+    volatile int* drain_flag = &drain_s;
+    float2* merge_s = reinterpret_cast<float2*>(smem + L_MERGE);
+    double* ll_s = reinterpret_cast<double*>(smem + L_MERGE);      // after the last tile
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int64_t ntiles = (p.n + WIDE_TILE - 1) / WIDE_TILE;
+    const int64_t ntl = ((int64_t)blockIdx.x < ntiles) ? (ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+    const int NC = p.NC, NZ = p.NZ;
+    const int NG = (NC + 3) >> 2;
+
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L_BAR);
+    auto BAR = [&](int i) { return smem_u32(&bars[i]); };
+    if (tid == 0) {
+        abort_s = 0;
+        drain_s = 0;
+        for (int s = 0; s < L_SLOTS; ++s) { bar_init(BAR(LB_FULL + s), 1); bar_init(BAR(LB_EMPTY + s), 1); }
+        bar_init(BAR(LB_LFULL), 1);
+        bar_init(BAR(LB_LEMPTY), 256);
+        bar_init(BAR(LB_FINAL), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == WT_MMA) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(512) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    fence_before();
+    __syncthreads();
+    fence_after();
+    const uint32_t tmem = tmem_base_s;
+
+    if (warp < 8) {
+        // =========================== softmax warps: thread = TMEM lane = point ===========================
+        // Warpgroup g reads chunks 2 g and 2 g + 1 of every group of four chunks; the two running (max, sum) pairs of a
+        // point are merged at the end of its tile.
+        const int grp = warp >> 2, wq = warp & 3;
+        const uint32_t lane_addr = ((uint32_t)(wq * 32)) << 16;
+        const int pt = wq * 32 + lane;                       // point within the tile
+        const double cref = *p.cref;
+        uint32_t uses = 0;
+        double ll_acc = 0.0;
+        for (int64_t i = 0; i < ntl; ++i) {
+            const int64_t row = (blockIdx.x + i * gridDim.x) * WIDE_TILE + pt;
+            float m_run = -1e30f, s_run = 0.f;               // finite start: blocks of -inf logits must not make NaN
+            for (int g = 0; g < NG; ++g) {
+                const int nch = (NC - 4 * g < 4) ? (NC - 4 * g) : 4;
+                const bool got = bar_wait(BAR(LB_LFULL), uses & 1u, abort_flag, p.status, false);
+                const bool ok = __all_sync(0xffffffffu, got);
+                fence_after();
+                ++uses;
+                if (ok) {
+#pragma unroll 1
+                    for (int cc = 0; cc < 2; ++cc) {
+                        const int c = 2 * grp + cc;
+                        if (c >= nch) break;                 // uniform over the warpgroup
+#pragma unroll 1
+                        for (int sub = 0; sub < 4; ++sub) {
+                            uint32_t v[32];
+                            tmem_ld32(tmem + c * 128 + sub * 32 + lane_addr, v);
+                            tmem_wait_ld();
+                            const int col0 = (4 * g + c) * 128 + sub * 32;
+                            const float4* tc4 = reinterpret_cast<const float4*>(p.tkck + col0);
+                            float l[32];
+                            float bmax = -CUDART_INF_F;
+#pragma unroll
+                            for (int j = 0; j < 32; j += 2) {
+                                const float4 q = __ldg(tc4 + (j >> 1));          // (t, c) of two components; same address in every lane
+                                l[j] = fmaf(__uint_as_float(v[j]), q.x, q.y);
+                                l[j + 1] = fmaf(__uint_as_float(v[j + 1]), q.z, q.w);
+                                bmax = fmaxf(bmax, fmaxf(l[j], l[j + 1]));
+                            }
+                            if (bmax > m_run) {
+                                s_run *= fast_ex2(m_run - bmax);
+                                m_run = bmax;
+                            }
+                            float acc0 = 0.f, acc1 = 0.f;
+#pragma unroll
+                            for (int j = 0; j < 32; j += 2) {
+                                acc0 += fast_ex2(l[j] - m_run);
+                                acc1 += fast_ex2(l[j + 1] - m_run);
+                            }
+                            s_run += acc0 + acc1;
+                        }
+                    }
+                }
+                fence_before();
+                bar_arrive(BAR(LB_LEMPTY));
+            }
+            // merge the two warpgroups' pairs; warpgroup 0 writes log2 Z
+            if (grp == 1) merge_s[pt] = make_float2(m_run, s_run);
+            named_bar_sync(1, 256);
+            if (grp == 0) {
+                const float2 o = merge_s[pt];
+                const float m = fmaxf(m_run, o.x);
+                const float s = s_run * fast_ex2(m_run - m) + o.y * fast_ex2(o.x - m);
+                if (row < p.n && !*abort_flag) {
+                    const double lz = cref + (double)m + (double)log2f(s);
+                    p.logz[row] = lz;
+                    ll_acc += lz;
+                }
+            }
+            named_bar_sync(2, 256);                          // merge_s is rewritten by the next tile
+        }
+        if (grp == 0) ll_s[pt] = ll_acc;
+        named_bar_sync(1, 256);
+        if (tid == 0) {
+            double s = 0.0;
+            for (int j = 0; j < 128; ++j) s += ll_s[j];
+            p.llpart[blockIdx.x] += s * 0.69314718055994530942;       // one owner per slot: launches add up
+        }
+    } else if (warp == WT_PRODUCER) {
+        // =========================== producer warp (TMA) ===========================
+        // Item order = order of use: per (tile, group, atom z) the tile's Y atom, then the group's coefficient atoms.
+        int64_t g = 0;
+        bool ok = true;
+        auto item = [&](const CUtensorMap* mh, const CUtensorMap* ml, int32_t row, int32_t z) -> bool {
+            const int slot = (int)(g % L_SLOTS);
+            const int64_t use = g / L_SLOTS;
+            if (use > 0) {
+                uint32_t w = 1;
+                if (lane == 0) w = bar_wait(BAR(LB_EMPTY + slot), (uint32_t)((use - 1) & 1), abort_flag, p.status, false) ? 1u : 0u;
+                if (!__shfl_sync(0xffffffffu, w, 0)) return false;
+            }
+            if (elect_one()) {
+                const uint32_t dst = smem_u32(smem + slot * SLOT);
+                bar_expect_tx(BAR(LB_FULL + slot), SLOT);
+                tma_load_3d(dst, mh, 0, row, z, BAR(LB_FULL + slot));
+                tma_load_3d(dst + SLOT / 2, ml, 0, row, z, BAR(LB_FULL + slot));
+            }
+            __syncwarp();
+            ++g;
+            return true;
+        };
+        for (int64_t i = 0; i < ntl && ok; ++i) {
+            const int32_t row0 = (int32_t)((blockIdx.x + i * gridDim.x) * WIDE_TILE);
+            for (int gq = 0; gq < NG && ok; ++gq) {
+                const int nch = (NC - 4 * gq < 4) ? (NC - 4 * gq) : 4;
+                for (int z = 0; z < NZ && ok; ++z) {
+                    ok = item(&tm_yhi, &tm_ylo, row0, z);
+                    for (int c = 0; c < nch && ok; ++c) ok = item(&tm_phi, &tm_plo, (4 * gq + c) * 128, z);
+                }
+            }
+        }
+        // the loads in flight must have landed before the CTA may exit, also after an abort
+        if (!ok || *abort_flag) {
+            for (int64_t h = (g > L_SLOTS ? g - L_SLOTS : 0); h < g; ++h) {
+                if (lane == 0) bar_wait(BAR(LB_FULL + (int)(h % L_SLOTS)), (uint32_t)((h / L_SLOTS) & 1), drain_flag, p.status, false);
+                __syncwarp();
+            }
+        }
+    } else {
+        // =========================== MMA warp ===========================
+        const uint32_t idesc = make_idesc(WIDE_TILE, 128, 0);
+        const uint64_t d0 = make_desc(smem_u32(smem), 16, 1024);
+        bool alive = true;
+        auto wait_all = [&](uint32_t bar, uint32_t parity) -> bool {
+            uint32_t ok = 1;
+            if (lane == 0) ok = bar_wait(bar, parity, abort_flag, p.status, false) ? 1u : 0u;
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            fence_after();
+            return ok != 0u;
+        };
+        int64_t g = 0;
+        uint32_t groups_done = 0;
+        for (int64_t i = 0; i < ntl && alive; ++i) {
+            for (int gq = 0; gq < NG && alive; ++gq) {
+                const int nch = (NC - 4 * gq < 4) ? (NC - 4 * gq) : 4;
+                if (groups_done > 0 && !wait_all(BAR(LB_LEMPTY), (groups_done - 1) & 1u)) { alive = false; break; }
+                for (int z = 0; z < NZ && alive; ++z) {
+                    const int sy = (int)(g % L_SLOTS);
+                    if (!wait_all(BAR(LB_FULL + sy), (uint32_t)((g / L_SLOTS) & 1))) { alive = false; break; }
+                    ++g;
+                    for (int c = 0; c < nch; ++c) {
+                        const int sp = (int)(g % L_SLOTS);
+                        if (!wait_all(BAR(LB_FULL + sp), (uint32_t)((g / L_SLOTS) & 1))) { alive = false; break; }
+                        ++g;
+                        if (elect_one()) {
+                            const uint64_t ah = d0 + ((sy * SLOT) >> 4), al = ah + ((SLOT / 2) >> 4);
+                            const uint64_t bh = d0 + ((sp * SLOT) >> 4), bl = bh + ((SLOT / 2) >> 4);
+                            const uint32_t d = tmem + c * 128;
+                            // the two small cross products of the atom first, then the leading one
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) mma_ss(d, ah + ((j * 32) >> 4), bl + ((j * 32) >> 4), idesc, (z > 0 || j > 0) ? 1u : 0u);
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) mma_ss(d, al + ((j * 32) >> 4), bh + ((j * 32) >> 4), idesc, 1u);
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) mma_ss(d, ah + ((j * 32) >> 4), bh + ((j * 32) >> 4), idesc, 1u);
+                            mma_commit(BAR(LB_EMPTY + sp));
+                            if (c == nch - 1) mma_commit(BAR(LB_EMPTY + sy));
+                            if (c == nch - 1 && z == NZ - 1) mma_commit(BAR(LB_LFULL));
+                        }
+                        __syncwarp();
+                    }
+                }
+                ++groups_done;
+            }
+        }
+        if (elect_one()) mma_commit(BAR(LB_FINAL));
+        __syncwarp();
+        if (lane == 0) bar_wait(BAR(LB_FINAL), 0, drain_flag, p.status, false);
+        __syncwarp();
+        fence_after();
+    }
+
+    fence_before();
+    __syncthreads();
+    if (warp == WT_MMA) {
+        fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512) : "memory");
+    }
+}
+
+// ------------------------------------------------------------------------------------------------------------------
+// Sweep 2
+constexpr int E_SLOTS = 6;
+constexpr int E_BAR = E_SLOTS * SLOT;
+constexpr int E_LZ = E_BAR + 256;                  // 2 x 256 floats: log2 Z - c_ref of the batch's points
+constexpr int E_SMEM = E_LZ + 2048 + 1024;
+enum { EB_FULL = 0, EB_EMPTY = E_SLOTS, EB_LFULL = 2 * E_SLOTS, EB_RREADY, EB_ACCFULL0, EB_ACCFULL1, EB_ACCFREE0,
+       EB_ACCFREE1, EB_FINAL, EB_COUNT };
+
+struct EmWideParams {
+    int64_t n;
+    int CL, R, NZ, pcols;
+    const float2* tkck;
+    const double* cref;
+    const double* logz;
+    float* partial;      // [R * CL][pcols][128]
+    int* status;
+};
+
+__global__ void __launch_bounds__(WT_THREADS, 1)
+em_wide_kernel(const EmWideParams p, const __grid_constant__ CUtensorMap tm_phi, const __grid_constant__ CUtensorMap tm_plo,
+               const __grid_constant__ CUtensorMap tm_ye_hi, const __grid_constant__ CUtensorMap tm_ye_lo,
+               const __grid_constant__ CUtensorMap tm_ym_hi, const __grid_constant__ CUtensorMap tm_ym_lo) {
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int abort_s, drain_s;
+    volatile int* abort_flag = &abort_s;
+    volatile int* drain_flag = &drain_s;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int slice = blockIdx.x % p.CL;                 // 128 components
+    const int range = blockIdx.x / p.CL;                 // takes batches range, range + R, ...
+    const int64_t nbatches = (p.n + WIDE_BATCH - 1) / WIDE_BATCH;
+    const int64_t nbl = (range < nbatches) ? (nbatches - range + p.R - 1) / p.R : 0;
+    const int NZ = p.NZ, NH = NZ >> 1;                   // atoms; half-slices of 64 dimensions (2 atoms = 128 columns)
+
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + E_BAR);
+    auto BAR = [&](int i) { return smem_u32(&bars[i]); };
+    if (tid == 0) {
+        abort_s = 0;
+        drain_s = 0;
+        for (int s = 0; s < E_SLOTS; ++s) { bar_init(BAR(EB_FULL + s), 1); bar_init(BAR(EB_EMPTY + s), 1); }
+        bar_init(BAR(EB_LFULL), 1);
+        bar_init(BAR(EB_RREADY), 256);
+        bar_init(BAR(EB_ACCFULL0), 1);  bar_init(BAR(EB_ACCFULL1), 1);
+        bar_init(BAR(EB_ACCFREE0), 256); bar_init(BAR(EB_ACCFREE1), 256);
+        bar_init(BAR(EB_FINAL), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == WT_MMA) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(512) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    fence_before();
+    __syncthreads();
+    fence_after();
+    const uint32_t tmem = tmem_base_s;
+    // TMEM columns: [0,128) / [128,256) the two alternating M-step accumulators (during the E-step: the accumulator of the
+    // two small cross products, points 0-255), [256,512) the main E-step product of the batch's 256 points, overwritten
+    // in place by the responsibilities: 32 points -> [r_hi 16 columns | r_lo 16 columns]
+    const uint32_t T_MAIN = tmem + 256;
+
+    if (warp < 8) {
+        // =========================== softmax / flush warps: thread = TMEM lane = component ===========================
+        const int grp = warp >> 2, wq = warp & 3;
+        const uint32_t lane_addr = ((uint32_t)(wq * 32)) << 16;
+        const int kloc = wq * 32 + lane;
+        const float2 tc = __ldg(p.tkck + slice * 128 + kloc);
+        const double cref = *p.cref;
+        float* lz_s = reinterpret_cast<float*>(smem + E_LZ);              // [2][256]
+        float* pblk = p.partial + (size_t)blockIdx.x * p.pcols * 128 + kloc;      // [column][component]: one owner per address
+        uint32_t acc_uses[2] = {0u, 0u};
+        for (int64_t b = 0; b < nbl; ++b) {
+            const int64_t row0 = (range + b * p.R) * WIDE_BATCH;
+            float* lz = lz_s + (b & 1) * 256;
+            {   // log2 Z - c_ref of the batch's points (+inf beyond n: those points get r = 0)
+                const int64_t row = row0 + (tid & 255);
+                lz[tid & 255] = (row < p.n) ? (float)(p.logz[row] - cref) : CUDART_INF_F;
+            }
+            named_bar_sync(1, 256);
+            const bool got = bar_wait(BAR(EB_LFULL), (uint32_t)(b & 1), abort_flag, p.status, false);
+            const bool ok = __all_sync(0xffffffffu, got);
+            fence_after();
+            float nsum = 0.f;
+            if (ok) {
+#pragma unroll 1
+                for (int ch = 0; ch < 4; ++ch) {
+                    const int p0 = 128 * grp + 32 * ch;                   // this thread's 32 points of the batch
+                    uint32_t vm[32], vc[32];
+                    tmem_ld32(T_MAIN + p0 + lane_addr, vm);
+                    tmem_ld32(tmem + p0 + lane_addr, vc);
+                    tmem_wait_ld();
+                    uint32_t hi[16], lo[16];
+#pragma unroll
+                    for (int j = 0; j < 32; j += 4) {
+                        const float4 z4 = *reinterpret_cast<const float4*>(lz + p0 + j);
+                        float r[4];
+                        const float zz[4] = {z4.x, z4.y, z4.z, z4.w};
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const float acc = __uint_as_float(vm[j + q]) + __uint_as_float(vc[j + q]);
+                            r[q] = fast_ex2(fmaf(acc, tc.x, tc.y - zz[q])) * RSCALE;
+                        }
+                        const __half2 h01 = __floats2half2_rn(r[0], r[1]), h23 = __floats2half2_rn(r[2], r[3]);
+                        const float2 b01 = __half22float2(h01), b23 = __half22float2(h23);
+                        const __half2 g01 = __floats2half2_rn(r[0] - b01.x, r[1] - b01.y), g23 = __floats2half2_rn(r[2] - b23.x, r[3] - b23.y);
+                        const float2 c01 = __half22float2(g01), c23 = __half22float2(g23);
+                        // N_k is the sum of exactly the weights the M-step uses (hi + lo)
+                        nsum += ((b01.x + c01.x) + (b01.y + c01.y)) + ((b23.x + c23.x) + (b23.y + c23.y));
+                        hi[j / 2] = *reinterpret_cast<const uint32_t*>(&h01);
+                        hi[j / 2 + 1] = *reinterpret_cast<const uint32_t*>(&h23);
+                        lo[j / 2] = *reinterpret_cast<const uint32_t*>(&g01);
+                        lo[j / 2 + 1] = *reinterpret_cast<const uint32_t*>(&g23);
+                    }
+                    tmem_st16(T_MAIN + p0 + lane_addr, hi);
+                    tmem_st16(T_MAIN + p0 + 16 + lane_addr, lo);
+                }
+                tmem_wait_st();
+            }
+            fence_before();
+            bar_arrive(BAR(EB_RREADY));
+            if (ok) atomicAdd(pblk + (size_t)(p.pcols - 2 + grp) * 128, nsum);         // N_k column of this warpgroup
+            // flush the M-step accumulators, half-slice by half-slice, as the MMA warp hands them over: warpgroup g takes
+            // columns [64 g, 64 g + 64) of the 128
+            for (int h = 0; h < NH; ++h) {
+                const int buf = h & 1;
+                const bool gotf = bar_wait(BAR(EB_ACCFULL0 + buf), acc_uses[buf] & 1u, abort_flag, p.status, false);
+                const bool okf = __all_sync(0xffffffffu, gotf);
+                ++acc_uses[buf];
+                fence_after();
+                if (okf) {
+#pragma unroll 1
+                    for (int c0 = 0; c0 < 64; c0 += 32) {
+                        uint32_t v[32];
+                        tmem_ld32(tmem + buf * 128 + grp * 64 + c0 + lane_addr, v);
+                        tmem_wait_ld();
+                        float* dst = pblk + (size_t)(h * 128 + grp * 64 + c0) * 128;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) atomicAdd(dst + (size_t)j * 128, __uint_as_float(v[j]));
+                    }
+                }
+                fence_before();
+                bar_arrive(BAR(EB_ACCFREE0 + buf));
+            }
+        }
+    } else if (warp == WT_PRODUCER) {
+        // =========================== producer warp (TMA) ===========================
+        // Items in order of use.  E-step, per atom z: the slice's coefficient atom (hi, lo: 2 x 16 KB in one slot), the batch's
+        // Y atom hi (256 points x 128 bytes: one slot), the same of the lo plane.  M-step, per half-slice and quarter of the
+        // batch: 64 points x 2 atoms of both planes (2 x 16 KB in one slot).
+        int64_t g = 0;
+        bool ok = true;
+        auto acquire = [&]() -> int {
+            const int slot = (int)(g % E_SLOTS);
+            const int64_t use = g / E_SLOTS;
+            if (use > 0) {
+                uint32_t w = 1;
+                if (lane == 0) w = bar_wait(BAR(EB_EMPTY + slot), (uint32_t)((use - 1) & 1), abort_flag, p.status, false) ? 1u : 0u;
+                if (!__shfl_sync(0xffffffffu, w, 0)) return -1;
+            }
+            return slot;
+        };
+        for (int64_t b = 0; b < nbl && ok; ++b) {
+            const int32_t row0 = (int32_t)((range + b * p.R) * WIDE_BATCH);
+            for (int z = 0; z < NZ && ok; ++z) {
+                int slot = acquire();
+                if (slot < 0) { ok = false; break; }
+                if (elect_one()) {
+                    const uint32_t dst = smem_u32(smem + slot * SLOT);
+                    bar_expect_tx(BAR(EB_FULL + slot), SLOT);
+                    tma_load_3d(dst, &tm_phi, 0, slice * 128, z, BAR(EB_FULL + slot));
+                    tma_load_3d(dst + SLOT / 2, &tm_plo, 0, slice * 128, z, BAR(EB_FULL + slot));
+                }
+                __syncwarp();
+                ++g;
+                for (int pl = 0; pl < 2 && ok; ++pl) {
+                    slot = acquire();
+                    if (slot < 0) { ok = false; break; }
+                    if (elect_one()) {
+                        bar_expect_tx(BAR(EB_FULL + slot), SLOT);
+                        tma_load_3d(smem_u32(smem + slot * SLOT), pl ? &tm_ye_lo : &tm_ye_hi, 0, row0, z, BAR(EB_FULL + slot));
+                    }
+                    __syncwarp();
+                    ++g;
+                }
+            }
+            for (int h = 0; h < NH && ok; ++h) {
+                for (int q4 = 0; q4 < 4 && ok; ++q4) {
+                    const int slot = acquire();
+                    if (slot < 0) { ok = false; break; }
+                    if (elect_one()) {
+                        const uint32_t dst = smem_u32(smem + slot * SLOT);
+                        bar_expect_tx(BAR(EB_FULL + slot), SLOT);
+                        tma_load_3d(dst, &tm_ym_hi, 0, row0 + 64 * q4, 2 * h, BAR(EB_FULL + slot));
+                        tma_load_3d(dst + SLOT / 2, &tm_ym_lo, 0, row0 + 64 * q4, 2 * h, BAR(EB_FULL + slot));
+                    }
+                    __syncwarp();
+                    ++g;
+                }
+            }
+        }
+        if (!ok || *abort_flag) {
+            for (int64_t h = (g > E_SLOTS ? g - E_SLOTS : 0); h < g; ++h) {
+                if (lane == 0) bar_wait(BAR(EB_FULL + (int)(h % E_SLOTS)), (uint32_t)((h / E_SLOTS) & 1), drain_flag, p.status, false);
+                __syncwarp();
+            }
+        }
+    } else {
+        // =========================== MMA warp ===========================
+        const uint32_t id_e = make_idesc(128, WIDE_BATCH, 0);       // E-step: M = 128 components, N = 256 points, both K-major
+        const uint32_t id_m = make_idesc(128, 128, 1);              // M-step: N = 128 statistics columns, B MN-major
+        const uint64_t dk = make_desc(smem_u32(smem), 16, 1024);    // K-major view of the ring
+        const uint64_t dm = make_desc(smem_u32(smem), 8192, 1024);  // MN-major view: 64-column atoms of 64 points, 8192 bytes apart
+        bool alive = true;
+        auto wait_all = [&](uint32_t bar, uint32_t parity) -> bool {
+            uint32_t ok = 1;
+            if (lane == 0) ok = bar_wait(bar, parity, abort_flag, p.status, false) ? 1u : 0u;
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            fence_after();
+            return ok != 0u;
+        };
+        int64_t g = 0;
+        uint32_t full_cnt[2] = {0u, 0u}, freed_cnt[2] = {0u, 0u};
+        // an accumulator may be written again only when every earlier hand-over of it has been flushed
+        auto ensure_free = [&](int buf) -> bool {
+            while (freed_cnt[buf] < full_cnt[buf]) {
+                if (!wait_all(BAR(EB_ACCFREE0 + buf), freed_cnt[buf] & 1u)) return false;
+                ++freed_cnt[buf];
+            }
+            return true;
+        };
+        for (int64_t b = 0; b < nbl && alive; ++b) {
+            // ---- E-step: the cross products use columns [0, 256), i.e. both M-step accumulators
+            if (!ensure_free(0) || !ensure_free(1)) { alive = false; break; }
+            for (int z = 0; z < NZ && alive; ++z) {
+                int sl[3];
+                for (int q = 0; q < 3; ++q) {
+                    sl[q] = (int)(g % E_SLOTS);
+                    if (!wait_all(BAR(EB_FULL + sl[q]), (uint32_t)((g / E_SLOTS) & 1))) { alive = false; break; }
+                    ++g;
+                }
+                if (!alive) break;
+                if (elect_one()) {
+                    const uint64_t ph = dk + ((sl[0] * SLOT) >> 4), plo = ph + ((SLOT / 2) >> 4);
+                    const uint64_t yh = dk + ((sl[1] * SLOT) >> 4), yl = dk + ((sl[2] * SLOT) >> 4);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) mma_ss(tmem, plo + ((j * 32) >> 4), yh + ((j * 32) >> 4), id_e, (z > 0 || j > 0) ? 1u : 0u);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) mma_ss(tmem, ph + ((j * 32) >> 4), yl + ((j * 32) >> 4), id_e, 1u);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) mma_ss(T_MAIN, ph + ((j * 32) >> 4), yh + ((j * 32) >> 4), id_e, (z > 0 || j > 0) ? 1u : 0u);
+                    mma_commit(BAR(EB_EMPTY + sl[0]));
+                    mma_commit(BAR(EB_EMPTY + sl[1]));
+                    mma_commit(BAR(EB_EMPTY + sl[2]));
+                    if (z == NZ - 1) mma_commit(BAR(EB_LFULL));
+                }
+                __syncwarp();
+            }
+            if (!alive) break;
+            // ---- M-step
+            if (!wait_all(BAR(EB_RREADY), (uint32_t)(b & 1))) { alive = false; break; }
+            for (int h = 0; h < NH && alive; ++h) {
+                const int buf = h & 1;
+                if (!ensure_free(buf)) { alive = false; break; }
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    const int s = (int)(g % E_SLOTS);
+                    if (!wait_all(BAR(EB_FULL + s), (uint32_t)((g / E_SLOTS) & 1))) { alive = false; break; }
+                    ++g;
+                    if (elect_one()) {
+                        const uint64_t yh = dm + ((s * SLOT) >> 4), yl = yh + ((SLOT / 2) >> 4);
+                        const uint32_t d = tmem + buf * 128;
+                        // A operand: 16 points per k-step; points 32 c .. 32 c + 31 sit in columns [32 c, 32 c + 16) (r_hi) and
+                        // [32 c + 16, 32 c + 32) (r_lo) of the main buffer
+#pragma unroll
+                        for (int ks = 0; ks < 4; ++ks) {
+                            const int kg = 4 * q4 + ks;
+                            mma_ts(d, T_MAIN + (kg >> 1) * 32 + (kg & 1) * 8, yh + ((ks * 2048) >> 4), id_m, (q4 > 0 || ks > 0) ? 1u : 0u);
+                        }
+#pragma unroll
+                        for (int ks = 0; ks < 4; ++ks) {
+                            const int kg = 4 * q4 + ks;
+                            mma_ts(d, T_MAIN + (kg >> 1) * 32 + (kg & 1) * 8, yl + ((ks * 2048) >> 4), id_m, 1u);
+                        }
+#pragma unroll
+                        for (int ks = 0; ks < 4; ++ks) {
+                            const int kg = 4 * q4 + ks;
+                            mma_ts(d, T_MAIN + (kg >> 1) * 32 + (kg & 1) * 8 + 16, yh + ((ks * 2048) >> 4), id_m, 1u);
+                        }
+                        mma_commit(BAR(EB_EMPTY + s));
+                        if (q4 == 3) mma_commit(BAR(EB_ACCFULL0 + buf));
+                    }
+                    __syncwarp();
+                }
+                if (alive) ++full_cnt[buf];
+            }
+        }
+        if (elect_one()) mma_commit(BAR(EB_FINAL));
+        __syncwarp();
+        if (lane == 0) bar_wait(BAR(EB_FINAL), 0, drain_flag, p.status, false);
+        __syncwarp();
+        fence_after();
+    }
+
+    fence_before();
+    __syncthreads();
+    if (warp == WT_MMA) {
+        fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512) : "memory");
+    }
+}
+
+// ------------------------------------------------------------------------------------------------------------------
+// X -> the two fp16 planes of Y = [u | u^2 + kap], u = s_d (x - g_d).  Row i of a plane holds 2 Dpad halves: k-step ks (8
+// dimensions) occupies halves [16 ks, 16 ks + 8) = u and [16 ks + 8, 16 ks + 16) = u^2 + kap.  One thread converts one
+// (point, k-step) unit and writes 32 contiguous bytes per plane.  Rows n .. rows_padded - 1 are written as zeros.
+__global__ void __launch_bounds__(256) wide_transform_kernel(const float* __restrict__ X, int64_t n, int64_t rows_padded, int D,
+                                                             int Dpad, const float* __restrict__ sd, const float* __restrict__ kap,
+                                                             const float* __restrict__ gd, unsigned char* __restrict__ yhi,
+                                                             unsigned char* __restrict__ ylo, int* __restrict__ status) {
+    const int upr = Dpad >> 3;                           // units per row
+    const int64_t units = rows_padded * upr;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    const bool vec_ok = (D % 4 == 0) && ((reinterpret_cast<uintptr_t>(X) & 15) == 0);
+    const size_t pitch = (size_t)Dpad * 4;               // bytes per row of a plane
+    bool bad = false;
+    for (int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; u < units; u += stride) {
+        const int64_t row = u / upr;
+        const int ks = (int)(u - row * upr), d0 = ks * 8;
+        const bool valid = row < n;
+        float x[8];
+        if (valid && vec_ok && d0 + 8 <= D) {
+            const float4 a = __ldg(reinterpret_cast<const float4*>(X + row * D + d0));
+            const float4 b = __ldg(reinterpret_cast<const float4*>(X + row * D + d0 + 4));
+            x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
+        } else {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) x[j] = (valid && d0 + j < D) ? __ldg(X + row * D + d0 + j) : 0.f;
+        }
+        uint32_t xh[4], xl[4], qh[4], ql[4];
+#pragma unroll
+        for (int j = 0; j < 8; j += 2) {
+            bad |= !(fabsf(x[j]) <= 3.0e38f) || !(fabsf(x[j + 1]) <= 3.0e38f);
+            const bool in0 = valid && d0 + j < D, in1 = valid && d0 + j + 1 < D;
+            float u0 = in0 ? (x[j] - __ldg(gd + d0 + j)) * __ldg(sd + d0 + j) : 0.f;
+            float u1 = in1 ? (x[j + 1] - __ldg(gd + d0 + j + 1)) * __ldg(sd + d0 + j + 1) : 0.f;
+            u0 = fminf(fmaxf(u0, -240.f), 240.f);
+            u1 = fminf(fmaxf(u1, -240.f), 240.f);
+            const float q0 = in0 ? fmaf(u0, u0, __ldg(kap + d0 + j)) : 0.f;
+            const float q1 = in1 ? fmaf(u1, u1, __ldg(kap + d0 + j + 1)) : 0.f;
+            const __half2 h = __floats2half2_rn(u0, u1);
+            const float2 hf = __half22float2(h);
+            const __half2 g2 = __floats2half2_rn(u0 - hf.x, u1 - hf.y);
+            const __half2 sq = __floats2half2_rn(q0, q1);
+            const float2 sf = __half22float2(sq);
+            const __half2 t2 = __floats2half2_rn(q0 - sf.x, q1 - sf.y);
+            xh[j / 2] = *reinterpret_cast<const uint32_t*>(&h);
+            xl[j / 2] = *reinterpret_cast<const uint32_t*>(&g2);
+            qh[j / 2] = *reinterpret_cast<const uint32_t*>(&sq);
+            ql[j / 2] = *reinterpret_cast<const uint32_t*>(&t2);
+        }
+        uint4* oh = reinterpret_cast<uint4*>(yhi + row * pitch + ks * 32);
+        uint4* ol = reinterpret_cast<uint4*>(ylo + row * pitch + ks * 32);
+        oh[0] = make_uint4(xh[0], xh[1], xh[2], xh[3]);
+        oh[1] = make_uint4(qh[0], qh[1], qh[2], qh[3]);
+        ol[0] = make_uint4(xl[0], xl[1], xl[2], xl[3]);
+        ol[1] = make_uint4(ql[0], ql[1], ql[2], ql[3]);
+    }
+    if (bad) atomicOr(status, ST_BAD_X);
+}
+
+// ------------------------------------------------------------------------------------------------------------------
+// Parameter preparation (float64 arithmetic on K * D elements).
+// One block per dimension: centre g_d = sum_k pi_k mu_kd / sum_k pi_k, scale s_d = 2^-round(log2 rms_d) with
+// rms_d^2 = sum_k pi_k ((mu_kd - g_d)^2 + var_kd), and kap_d = s_d^2 sum_k pi_k ((mu_kd - g_d)^2 - var_kd): with that
+// constant a component's own points (x = mu + sigma z) give the term a u + b (u^2 + kap) of dimension d the expectation
+// w (mu'^2 - var) / 2 - w kap / (2 s^2), which vanishes on average over the mixture, so the contraction's partial sums are a
+// zero-mean walk over the dimensions instead of growing like D / 2.
+__global__ void __launch_bounds__(128) wide_scale_kernel(int D, int K, const float* __restrict__ pi, const float* __restrict__ mu,
+                                                         const float* __restrict__ var, float* __restrict__ sd,
+                                                         float* __restrict__ kap, float* __restrict__ gd) {
+    const int d = blockIdx.x, t = threadIdx.x;
+    __shared__ double r_a[128], r_b[128], r_w[128];
+    __shared__ double g_s;
+    double a = 0.0, w = 0.0;
+    if (d < D)
+        for (int k = t; k < K; k += 128) {
+            const double pk = (double)pi[k];
+            a += pk * (double)mu[(size_t)k * D + d];
+            w += pk;
+        }
+    r_a[t] = a; r_w[t] = w;
+    __syncthreads();
+    for (int o = 64; o > 0; o >>= 1) {
+        if (t < o) { r_a[t] += r_a[t + o]; r_w[t] += r_w[t + o]; }
+        __syncthreads();
+    }
+    if (t == 0) {
+        const float gf = (r_w[0] > 0.0) ? (float)(r_a[0] / r_w[0]) : 0.f;
+        g_s = (d < D && isfinite(gf)) ? (double)gf : 0.0;
+    }
+    __syncthreads();
+    const double g = g_s;
+    double m2 = 0.0, v = 0.0;
+    w = 0.0;
+    if (d < D)
+        for (int k = t; k < K; k += 128) {
+            const double pk = (double)pi[k];
+            const double m = (double)mu[(size_t)k * D + d] - g;
+            m2 += pk * m * m;
+            v += pk * (double)var[(size_t)k * D + d];
+            w += pk;
+        }
+    __syncthreads();
+    r_a[t] = m2; r_b[t] = v; r_w[t] = w;
+    __syncthreads();
+    for (int o = 64; o > 0; o >>= 1) {
+        if (t < o) { r_a[t] += r_a[t + o]; r_b[t] += r_b[t + o]; r_w[t] += r_w[t + o]; }
+        __syncthreads();
+    }
+    if (t == 0) {
+        float s = 1.f, kp = 0.f;
+        double mm = r_a[0], vv = r_b[0];
+        if (r_w[0] > 0.0) { mm /= r_w[0]; vv /= r_w[0]; }
+        const double ms = mm + vv;
+        if (d < D && ms > 0.0 && isfinite(ms)) {
+            const double e = rint(0.5 * log2(ms));
+            s = (float)exp2(-fmin(fmax(e, -60.0), 60.0));
+            kp = (float)((mm - vv) * (double)s * (double)s);
+        }
+        sd[d] = s;
+        kap[d] = kp;
+        gd[d] = (float)g;
+    }
+}
+
+// One block per padded component: coefficient planes, t_k, c_k (float64), conditioning flag.
+__global__ void __launch_bounds__(256) wide_prepare_kernel(int D, int Dpad, int K, const float* __restrict__ pi,
+                                                           const float* __restrict__ mu, const float* __restrict__ var,
+                                                           const float* __restrict__ sd, const float* __restrict__ kap,
+                                                           const float* __restrict__ gd, __half* __restrict__ p_hi,
+                                                           __half* __restrict__ p_lo, float* __restrict__ tk,
+                                                           double* __restrict__ ckd, float* __restrict__ illb,
+                                                           float cond_limit, int* __restrict__ flags) {
+    extern __shared__ double ab_s[];                     // [2][Dpad]: a, b of this component
+    __shared__ double red[4][256];
+    const int k = blockIdx.x, t = threadIdx.x;
+    double mx = 0.0, csum = 0.0, cond2 = 0.0;
+    for (int d = t; d < Dpad; d += 256) {
+        double a = 0.0, b = 0.0;
+        if (k < K && d < D) {
+            const double v = (double)var[(size_t)k * D + d], m = (double)mu[(size_t)k * D + d] - (double)gd[d], s = (double)sd[d];
+            const double w = 1.4426950408889634074 / v;
+            a = w * m / s;
+            b = -0.5 * w / (s * s);
+            csum += m * m / v + log(6.283185307179586476925286766559 * v);
+            const double tau = 0.5 * w * 3.0 * (m * m + 9.0 * v);       // size of the dimension's terms at 3 sigma
+            cond2 += tau * tau;
+            mx = fmax(mx, fmax(fabs(a), fabs(b)));
+        }
+        ab_s[d] = a;
+        ab_s[Dpad + d] = b;
+    }
+    red[0][t] = mx; red[1][t] = csum; red[2][t] = cond2;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) {
+        if (t < o) {
+            red[0][t] = fmax(red[0][t], red[0][t + o]);
+            red[1][t] += red[1][t + o];
+            red[2][t] += red[2][t + o];
+        }
+        __syncthreads();
+    }
+    mx = red[0][0];
+    double tt = 1.0;
+    if (mx > 0.0 && isfinite(mx)) tt = exp2(floor(log2(mx)) - 9.0);      // max |P / t| in [512, 1024)
+    double ksum = 0.0;
+    __half* rh = p_hi + (size_t)k * 2 * Dpad;
+    __half* rl = p_lo + (size_t)k * 2 * Dpad;
+    for (int d = t; d < Dpad; d += 256) {
+        const double as = ab_s[d] / tt, bs = ab_s[Dpad + d] / tt;
+        const __half ah = __double2half(as), bh = __double2half(bs);
+        const __half al = __double2half(as - (double)__half2float(ah)), bl = __double2half(bs - (double)__half2float(bh));
+        const int cx = 16 * (d >> 3) + (d & 7);          // k-step interleaved column order, slices of 128 dimensions in sequence
+        rh[cx] = ah; rh[cx + 8] = bh; rl[cx] = al; rl[cx + 8] = bl;
+        // what the contraction adds through the shifted squares is taken out of c_k
+        ksum += tt * ((double)__half2float(bh) + (double)__half2float(bl)) * (double)kap[d];
+    }
+    __syncthreads();
+    red[3][t] = ksum;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) {
+        if (t < o) red[3][t] += red[3][t + o];
+        __syncthreads();
+    }
+    if (t == 0) {
+        double c = -CUDART_INF;
+        if (k < K) {
+            const float pk = pi[k];
+            if (pk > 0.f) c = 1.4426950408889634074 * (log((double)pk) - 0.5 * red[1][0]) - red[3][0];
+        }
+        // error estimate of the approximate log2 z: operand rounding at 2^-22 of every term, terms of independent sign
+        const double est = 4.0 * 2.384185791015625e-07 * sqrt(red[2][0]);
+        float margin = 0.f;
+        if (k < K && !(est <= (double)cond_limit)) {
+            margin = (float)fmin(8.0 * est, 1e30);
+            if (!(margin > 0.f)) margin = 1e30f;
+            atomicOr(flags, 1);
+            atomicAdd(flags + 4, 1);
+        }
+        tk[k] = (float)tt;
+        ckd[k] = c;
+        illb[k] = margin;
+    }
+}
+
+// c_ref = the largest finite c_k; tkck[k] = (t_k, c_k - c_ref) in fp32 (-inf where the component takes no part).
+__global__ void __launch_bounds__(1024) wide_cref_kernel(int Kpad, const float* __restrict__ tk, const double* __restrict__ ckd,
+                                                         const float* __restrict__ illb, double* __restrict__ cref,
+                                                         float2* __restrict__ tkck) {
+    __shared__ double red[1024];
+    double m = -CUDART_INF;
+    for (int k = threadIdx.x; k < Kpad; k += 1024)
+        if (!(illb[k] > 0.f) && isfinite(ckd[k])) m = fmax(m, ckd[k]);
+    red[threadIdx.x] = m;
+    __syncthreads();
+    for (int o = 512; o > 0; o >>= 1) {
+        if (threadIdx.x < o) red[threadIdx.x] = fmax(red[threadIdx.x], red[threadIdx.x + o]);
+        __syncthreads();
+    }
+    const double r = isfinite(red[0]) ? red[0] : 0.0;
+    if (threadIdx.x == 0) *cref = r;
+    for (int k = threadIdx.x; k < Kpad; k += 1024) {
+        const bool in = !(illb[k] > 0.f) && isfinite(ckd[k]);
+        tkck[k] = make_float2(tk[k], in ? (float)(ckd[k] - r) : -CUDART_INF_F);
+    }
+}
+
+// stats += sum over the R partial blocks of a component slice (fixed order, float64), undoing the responsibility scale,
+// the per-dimension scale and centre, and the column order; the partial blocks are left as they are (the caller clears them).
+__global__ void wide_reduce_kernel(int D, int K, int CL, int R, int pcols, const float* __restrict__ partial,
+                                   const float* __restrict__ sd, const float* __restrict__ kap, const float* __restrict__ gd,
+                                   double* __restrict__ Nk, double* __restrict__ S1, double* __restrict__ S2) {
+    const size_t KD = (size_t)K * D, per = (size_t)K + 2 * KD;
+    const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= per) return;
+    const double unscale = 1.0 / (double)TC_RSCALE;
+    auto column = [&](int col, int k) {
+        double s = 0.0;
+        const int sl = k >> 7, kl = k & 127;
+        for (int q = 0; q < R; ++q) s += (double)partial[((size_t)(q * CL + sl) * pcols + col) * 128 + kl];
+        return s;
+    };
+    if (e < (size_t)K) {
+        const int k = (int)e;
+        Nk[e] += (column(pcols - 2, k) + column(pcols - 1, k)) * unscale;
+        return;
+    }
+    const bool second = e >= K + KD;
+    const size_t j = second ? (e - K - KD) : (e - K);
+    const int k = (int)(j / D), d = (int)(j % D);
+    const int col = 16 * (d >> 3) + (d & 7);
+    const double s_d = (double)sd[d], g = (double)gd[d];
+    const double nk_raw = column(pcols - 2, k) + column(pcols - 1, k);
+    const double nk = nk_raw * unscale;
+    const double s1c = column(col, k) * unscale / s_d;
+    if (!second) {
+        S1[j] += s1c + g * nk;
+    } else {
+        const double s2c = (column(col + 8, k) - (double)kap[d] * nk_raw) * unscale / (s_d * s_d);
+        S2[j] += s2c + 2.0 * g * s1c + g * g * nk;
+    }
+}
+
+// A plane [rows][pitch bytes] seen as a 3-D tensor (x = 64 halves of an atom's row, y = row, z = atom): a box of
+// (64, box_rows, box_atoms) lands in shared memory as [atom][row][128 bytes], each 128-byte row swizzled.
+cudaError_t wide_make_map(CUtensorMap* tm, void* base, int64_t rows, int64_t pitch, int atoms, int box_rows, int box_atoms) {
+    const cuuint64_t dims[3] = {64, (cuuint64_t)rows, (cuuint64_t)atoms};
+    const cuuint64_t strides[2] = {(cuuint64_t)pitch, 128};
+    const cuuint32_t box[3] = {64, (cuuint32_t)box_rows, (cuuint32_t)box_atoms};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    typedef CUresult (*encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    static encode_fn encode = nullptr;
+    if (!encode) {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        const cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
+        if (e != cudaSuccess) return e;
+        if (q != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
+        encode = reinterpret_cast<encode_fn>(fn);
+    }
+    const CUresult r = encode(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, base, dims, strides, box, estr,
+                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+inline int64_t rows_padded_of(int64_t n) { return (n + WIDE_BATCH - 1) / WIDE_BATCH * WIDE_BATCH; }
+
+}  // namespace
+
+bool wide_supports(int D, int K) { return D > 128 && D <= WIDE_MAX_D && K >= 1 && K <= WIDE_MAX_K; }
+
+WidePlan wide_plan(int D, int K, int num_sms) {
+    WidePlan pl;
+    pl.n_slices = (D + 127) / 128;
+    pl.Dpad = pl.n_slices * 128;
+    pl.CL = (K + 127) / 128;
+    pl.Kpad = pl.CL * 128;
+    pl.R = num_sms / pl.CL;
+    if (pl.R < 1) pl.R = 1;
+    pl.pcols = 2 * pl.Dpad + 2;
+    return pl;
+}
+
+cudaError_t launch_prepare_wide(cudaStream_t s, int D, int K, const float* pi, const float* mu, const float* var,
+                                const WideBuffers& wb, float cond_limit) {
+    const WidePlan pl = wide_plan(D, K, 148);
+    cudaError_t e = cudaMemsetAsync(wb.flags, 0, 8 * sizeof(int), s);
+    if (e != cudaSuccess) return e;
+    wide_scale_kernel<<<pl.Dpad, 128, 0, s>>>(D, K, pi, mu, var, wb.sd, wb.kap, wb.gd);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    wide_prepare_kernel<<<pl.Kpad, 256, (size_t)2 * pl.Dpad * sizeof(double), s>>>(
+        D, pl.Dpad, K, pi, mu, var, wb.sd, wb.kap, wb.gd, reinterpret_cast<__half*>(wb.p_hi), reinterpret_cast<__half*>(wb.p_lo),
+        wb.tk, wb.ckd, wb.illb, cond_limit, wb.flags);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    wide_cref_kernel<<<1, 1024, 0, s>>>(pl.Kpad, wb.tk, wb.ckd, wb.illb, wb.cref, reinterpret_cast<float2*>(wb.tkck));
+    return cudaGetLastError();
+}
+
+cudaError_t launch_transform_wide(cudaStream_t s, const float* X, int64_t n, int D, const WideBuffers& wb, int* status) {
+    if (n < 1 || n > WIDE_PIECE) return cudaErrorInvalidValue;
+    const WidePlan pl = wide_plan(D, 1, 148);
+    const int64_t rp = rows_padded_of(n);
+    const int64_t units = rp * (pl.Dpad >> 3);
+    int64_t blocks = (units + 255) / 256;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    wide_transform_kernel<<<(unsigned)blocks, 256, 0, s>>>(X, n, rp, D, pl.Dpad, wb.sd, wb.kap, wb.gd, wb.y_hi, wb.y_lo, status);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_lse_wide(cudaStream_t s, int64_t n, int D, int K, const WideBuffers& wb, int num_sms, int* status) {
+    if (n < 1 || n > WIDE_PIECE) return cudaErrorInvalidValue;
+    const WidePlan pl = wide_plan(D, K, num_sms);
+    const int64_t rp = rows_padded_of(n);
+    const int64_t pitch = (int64_t)pl.Dpad * 4;
+    const int atoms = 4 * pl.n_slices;
+    CUtensorMap tm_yhi, tm_ylo, tm_phi, tm_plo;
+    cudaError_t e = wide_make_map(&tm_yhi, wb.y_hi, rp, pitch, atoms, WIDE_TILE, 1);
+    if (e == cudaSuccess) e = wide_make_map(&tm_ylo, wb.y_lo, rp, pitch, atoms, WIDE_TILE, 1);
+    if (e == cudaSuccess) e = wide_make_map(&tm_phi, wb.p_hi, pl.Kpad, pitch, atoms, 128, 1);
+    if (e == cudaSuccess) e = wide_make_map(&tm_plo, wb.p_lo, pl.Kpad, pitch, atoms, 128, 1);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(lse_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L_SMEM);
+    if (e != cudaSuccess) return e;
+    LseParams p;
+    p.n = n; p.NC = pl.CL; p.NZ = atoms;
+    p.tkck = reinterpret_cast<const float2*>(wb.tkck); p.cref = wb.cref; p.logz = wb.logz; p.llpart = wb.llpart; p.status = status;
+    const int64_t ntiles = (n + WIDE_TILE - 1) / WIDE_TILE;
+    const unsigned grid = (unsigned)(ntiles < num_sms ? ntiles : num_sms);
+    lse_wide_kernel<<<grid, WT_THREADS, L_SMEM, s>>>(p, tm_yhi, tm_ylo, tm_phi, tm_plo);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_em_wide(cudaStream_t s, int64_t n, int D, int K, const WideBuffers& wb, int num_sms, int* status) {
+    if (n < 1 || n > WIDE_PIECE) return cudaErrorInvalidValue;
+    const WidePlan pl = wide_plan(D, K, num_sms);
+    const int64_t rp = rows_padded_of(n);
+    const int64_t pitch = (int64_t)pl.Dpad * 4;
+    const int atoms = 4 * pl.n_slices;
+    CUtensorMap tm_phi, tm_plo, tm_ye_hi, tm_ye_lo, tm_ym_hi, tm_ym_lo;
+    cudaError_t e = wide_make_map(&tm_phi, wb.p_hi, pl.Kpad, pitch, atoms, 128, 1);
+    if (e == cudaSuccess) e = wide_make_map(&tm_plo, wb.p_lo, pl.Kpad, pitch, atoms, 128, 1);
+    if (e == cudaSuccess) e = wide_make_map(&tm_ye_hi, wb.y_hi, rp, pitch, atoms, WIDE_BATCH, 1);
+    if (e == cudaSuccess) e = wide_make_map(&tm_ye_lo, wb.y_lo, rp, pitch, atoms, WIDE_BATCH, 1);
+    if (e == cudaSuccess) e = wide_make_map(&tm_ym_hi, wb.y_hi, rp, pitch, atoms, 64, 2);
+    if (e == cudaSuccess) e = wide_make_map(&tm_ym_lo, wb.y_lo, rp, pitch, atoms, 64, 2);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(em_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, E_SMEM);
+    if (e != cudaSuccess) return e;
+    EmWideParams p;
+    p.n = n; p.CL = pl.CL; p.R = pl.R; p.NZ = atoms; p.pcols = pl.pcols;
+    p.tkck = reinterpret_cast<const float2*>(wb.tkck); p.cref = wb.cref; p.logz = wb.logz; p.partial = wb.partial; p.status = status;
+    em_wide_kernel<<<(unsigned)(pl.CL * pl.R), WT_THREADS, E_SMEM, s>>>(p, tm_phi, tm_plo, tm_ye_hi, tm_ye_lo, tm_ym_hi, tm_ym_lo);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_reduce_wide(cudaStream_t s, int D, int K, const WideBuffers& wb, int num_sms, double* Nk, double* S1,
+                               double* S2) {
+    const WidePlan pl = wide_plan(D, K, num_sms);
+    const size_t per = (size_t)K + 2 * (size_t)K * D;
+    wide_reduce_kernel<<<(unsigned)((per + 255) / 256), 256, 0, s>>>(D, K, pl.CL, pl.R, pl.pcols, wb.partial, wb.sd, wb.kap, wb.gd, Nk, S1, S2);
+    return cudaGetLastError();
+}
+
+}  // namespace fg

@@ -2,6 +2,7 @@
 // host-streaming variant.  Every step of the numerical path runs in the CUDA kernels of the other files.
 #include "internal.cuh"
 #include "em_tc.cuh"
+#include "em_wide.cuh"
 
 #include <algorithm>
 #include <cmath>
@@ -32,6 +33,10 @@ struct ScratchLayout {
     size_t w2, c2, c2d, center, partials, logZ2, llpart, result, stats, total;
     size_t tc_phi, tc_plo, tc_tk, tc_ck, tc_sd, tc_kap, tc_gd, tc_illb, tc_flags, tc_xg, tc_xl, tc_partial, tc_llpart, tc_partial_bytes, tc_yhi, tc_ylo, tc_phirm, tc_plorm, tc_tkck, tc_illlist, tc_illcache, tc_decdim, tc_decw, tc_decmu;
     bool tc;
+    // the tensor-core path for D > 128
+    size_t w_sd, w_kap, w_gd, w_phi, w_plo, w_tk, w_tkck, w_ckd, w_cref, w_illb, w_flags, w_yhi, w_ylo, w_logz, w_partial, w_llpart;
+    size_t w_partial_bytes;
+    bool wide;
 };
 
 // planes: include the fp16 planes of Y (tensor path only; 2 x TC_YPLANE_BYTES, placed last so that no other offset moves)
@@ -83,6 +88,29 @@ ScratchLayout scratch_layout(int D, int K, bool planes) {
         L.tc_yhi = take(TC_YPLANE_BYTES);
         L.tc_ylo = take(TC_YPLANE_BYTES);
     }
+    L.w_sd = L.w_kap = L.w_gd = L.w_phi = L.w_plo = L.w_tk = L.w_tkck = L.w_ckd = L.w_cref = L.w_illb = L.w_flags = L.w_yhi = L.w_ylo = L.w_logz = L.w_partial = L.w_llpart = 0;
+    L.w_partial_bytes = 0;
+    L.wide = wide_supports(D, K) && planes;
+    if (L.wide) {
+        const WidePlan wp = wide_plan(D, K, 160);
+        L.w_sd = take((size_t)wp.Dpad * 4);
+        L.w_kap = take((size_t)wp.Dpad * 4);
+        L.w_gd = take((size_t)wp.Dpad * 4);
+        L.w_phi = take((size_t)wp.Kpad * wp.Dpad * 4);
+        L.w_plo = take((size_t)wp.Kpad * wp.Dpad * 4);
+        L.w_tk = take((size_t)wp.Kpad * 4);
+        L.w_tkck = take((size_t)wp.Kpad * 8);
+        L.w_ckd = take((size_t)wp.Kpad * 8);
+        L.w_cref = take(8);
+        L.w_illb = take((size_t)wp.Kpad * 4);
+        L.w_flags = take(32);
+        L.w_logz = take((size_t)WIDE_PIECE * 8);
+        L.w_partial_bytes = (size_t)wp.R * wp.CL * wp.pcols * 128 * 4;
+        L.w_partial = take(L.w_partial_bytes);
+        L.w_llpart = take(256 * 8);
+        L.w_yhi = take((size_t)WIDE_PIECE * wp.Dpad * 4);
+        L.w_ylo = take((size_t)WIDE_PIECE * wp.Dpad * 4);
+    }
     L.total = off;
     return L;
 }
@@ -116,6 +144,8 @@ struct gmm_ctx {
     float tc_cond_scale = 1.5e-4f;
     int tc_flush = TC_FLUSH;
     int64_t tc_piece = TC_YPOINTS;   // points per launch of the tile kernel (<= capacity of the Y planes)
+    int64_t wide_piece = WIDE_PIECE; // points per pair of sweeps of the D > 128 tensor path
+    int sms = 148;                   // multiprocessors of the device
     int tc_n_ill = 0;                // ill-conditioned components at the last result that was read back (picks the filter)
     int tc_force_filter = -1;        // GMM_TC_FILTER=plain / tight: 0 / 1 (tests); -1: automatic
     int sticky_status = 0;           // status bits read off the device but not yet reported (see ensure_scratch)
@@ -171,6 +201,26 @@ struct gmm_ctx {
         b.dec_mu = reinterpret_cast<float*>(scratch + lay.tc_decmu);
         return b;
     }
+    WideBuffers wide() const {
+        WideBuffers b;
+        b.sd = reinterpret_cast<float*>(scratch + lay.w_sd);
+        b.kap = reinterpret_cast<float*>(scratch + lay.w_kap);
+        b.gd = reinterpret_cast<float*>(scratch + lay.w_gd);
+        b.p_hi = scratch + lay.w_phi;
+        b.p_lo = scratch + lay.w_plo;
+        b.tk = reinterpret_cast<float*>(scratch + lay.w_tk);
+        b.tkck = reinterpret_cast<float*>(scratch + lay.w_tkck);
+        b.ckd = reinterpret_cast<double*>(scratch + lay.w_ckd);
+        b.cref = reinterpret_cast<double*>(scratch + lay.w_cref);
+        b.illb = reinterpret_cast<float*>(scratch + lay.w_illb);
+        b.flags = reinterpret_cast<int*>(scratch + lay.w_flags);
+        b.y_hi = scratch + lay.w_yhi;
+        b.y_lo = scratch + lay.w_ylo;
+        b.logz = reinterpret_cast<double*>(scratch + lay.w_logz);
+        b.partial = reinterpret_cast<float*>(scratch + lay.w_partial);
+        b.llpart = reinterpret_cast<double*>(scratch + lay.w_llpart);
+        return b;
+    }
 };
 
 namespace {
@@ -203,10 +253,15 @@ int fail(gmm_ctx* ctx, int code, const char* fmt, ...) {
 // The tensor path runs when it is forced or when AUTO picks it for the shape: only then are the planes of Y needed.
 bool auto_is_tensor(int D, int K) { return tc_supports(D, K) && K >= 64 && D >= 8; }
 // AUTO also uses the tensor-core assignment for the larger K that only the assignment kernels take: planes are needed then
-bool auto_wants_planes(int D, int K) { return tc_assign_supports(D, K) && K >= 64 && D >= 8; }
+// (and for D > 128 the two-sweep tensor path, which needs its own planes)
+bool auto_wants_planes(int D, int K) { return (tc_assign_supports(D, K) && K >= 64 && D >= 8) || (wide_supports(D, K) && K >= 64); }
+// Points per component from which AUTO takes the tensor path for D > 128: its logits carry an error of about 1e-4 in the
+// log2 domain (fp32 accumulators of magnitude ~100), which the averaging over a component's points must absorb.
+constexpr int64_t WIDE_AUTO_MIN_POINTS_PER_COMPONENT = 32;
 
 int ensure_scratch(gmm_ctx* ctx, int D, int K) {
-    const bool planes = tc_assign_supports(D, K) && (ctx->path == GMM_PATH_TENSOR || (ctx->path == GMM_PATH_AUTO && auto_wants_planes(D, K)));
+    const bool planes = (tc_assign_supports(D, K) || wide_supports(D, K)) &&
+                        (ctx->path == GMM_PATH_TENSOR || (ctx->path == GMM_PATH_AUTO && auto_wants_planes(D, K)));
     if (ctx->scratch && D == ctx->capD && K == ctx->capK && planes == ctx->capPlanes) return GMM_OK;
     const ScratchLayout L = scratch_layout(D, K, planes);
     if (ctx->scratch) {
@@ -237,6 +292,7 @@ int ensure_scratch(gmm_ctx* ctx, int D, int K) {
     ctx->capPlanes = planes;
     CU(cudaMemsetAsync(ctx->result(), 0, sizeof(DevResult), ctx->stream));
     ctx->tc_Q = 0;
+    CU(cudaDeviceGetAttribute(&ctx->sms, cudaDevAttrMultiProcessorCount, ctx->device));
     if (L.tc && tc_supports(D, K)) {
         int q = 0;
         CU(tc_max_clusters(D, K, &q));
@@ -302,10 +358,29 @@ int prepare_and_choose(gmm_ctx* ctx, int64_t N, int D, int K, const float* pi, c
                        int* path) {
     KL(launch_prepare_fp32(ctx->stream, D, K, pi, mu, var, ctx->w2(), ctx->c2(), ctx->c2d(), ctx->center(), &ctx->result()->status));
     if ((size_t)K * D > ((size_t)1 << 12)) ctx->launches++;      // but for tiny problems, the centre of the means is a launch of its own
+    if (wide_supports(D, K)) {
+        // D > 128: the two-sweep tensor path when forced, or under AUTO from enough points per component on; parameter sets
+        // in which the preparation flags an ill-conditioned component go to the FP32 kernels (read back: one small
+        // synchronisation per step, against seconds of compute at these shapes).
+        const bool want = ctx->lay.wide && (ctx->path == GMM_PATH_TENSOR ||
+                                            (ctx->path == GMM_PATH_AUTO && K >= 64 && N >= WIDE_AUTO_MIN_POINTS_PER_COMPONENT * K));
+        *path = GMM_PATH_FP32;
+        if (!want) return GMM_OK;
+        float limit = ctx->tc_cond_limit;
+        if (limit < 0.f) limit = ctx->tc_cond_scale * std::sqrt((float)((double)N / (double)K));
+        const WideBuffers wb = ctx->wide();
+        KL(launch_prepare_wide(ctx->stream, D, K, pi, mu, var, wb, limit));
+        ctx->launches += 2;
+        int n_ill = 0;
+        CU(cudaMemcpyAsync(&n_ill, wb.flags + 4, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
+        CU(cudaStreamSynchronize(ctx->stream));
+        if (n_ill == 0) *path = GMM_PATH_TENSOR;
+        return GMM_OK;
+    }
     const bool tc_ok = ctx->lay.tc && ctx->tc_Q >= 1;
     const bool tc_auto = tc_ok && gmm_auto_path(D, K) == GMM_PATH_TENSOR;
     if (ctx->path == GMM_PATH_TENSOR && !tc_ok)
-        return fail(ctx, GMM_EUNSUPPORTED, "the tensor-core path needs D <= 128 and K <= 4096 (got D=%d K=%d)", D, K);
+        return fail(ctx, GMM_EUNSUPPORTED, "the tensor-core path needs D <= %d and K <= 4096 (got D=%d K=%d)", WIDE_MAX_D, D, K);
     if (ctx->path == GMM_PATH_FP32 || !tc_ok || (ctx->path == GMM_PATH_AUTO && !tc_auto)) {
         *path = GMM_PATH_FP32;
         return GMM_OK;
@@ -330,6 +405,26 @@ int prepare_and_choose(gmm_ctx* ctx, int64_t N, int D, int K, const float* pi, c
 // Adds the statistics of n device-resident points to (Nk, S1, S2) and their log-likelihood to result()->ll[slot].
 int accumulate_points(gmm_ctx* ctx, int path, const float* X, int64_t n, int D, int K, const float* mu, double* Nk,
                       double* S1, double* S2, int slot) {
+    if (path == GMM_PATH_TENSOR && wide_supports(D, K)) {
+        // Two sweeps per piece of at most 2^17 points (the capacity of the planes of Y and of the log2 Z buffer): planes,
+        // log-sum-exp, responsibilities + statistics into per-CTA fp32 partials, which are folded into the float64
+        // statistics piece by piece (no fp32 chain longer than a piece's batches).
+        const WideBuffers wb = ctx->wide();
+        const int grid1 = ctx->sms;
+        CU(cudaMemsetAsync(wb.llpart, 0, 256 * 8, ctx->stream));
+        for (int64_t off = 0; off < n; off += ctx->wide_piece) {
+            const int64_t cnt = (n - off < ctx->wide_piece) ? (n - off) : ctx->wide_piece;
+            CU(cudaMemsetAsync(wb.partial, 0, ctx->lay.w_partial_bytes, ctx->stream));
+            CHECK(prof_begin(ctx));
+            KL(launch_transform_wide(ctx->stream, X + off * D, cnt, D, wb, &ctx->result()->status));
+            KL(launch_lse_wide(ctx->stream, cnt, D, K, wb, grid1, &ctx->result()->status));
+            KL(launch_em_wide(ctx->stream, cnt, D, K, wb, ctx->sms, &ctx->result()->status));
+            CHECK(prof_end(ctx));
+            KL(launch_reduce_wide(ctx->stream, D, K, wb, ctx->sms, Nk, S1, S2));
+        }
+        KL(launch_reduce_ll(ctx->stream, wb.llpart, grid1 < 256 ? grid1 : 256, &ctx->result()->ll[slot], true));
+        return GMM_OK;
+    }
     if (path == GMM_PATH_TENSOR) {
         const TcBuffers tb = ctx->tc();
         const TcPlan pl = tc_plan(D, K, 160);
@@ -438,6 +533,10 @@ int gmm_create(gmm_ctx** out, int device, void* cuda_stream) {
     if (const char* e = std::getenv("GMM_TC_COND_LIMIT")) ctx->tc_cond_limit = (float)std::atof(e);
     if (const char* e = std::getenv("GMM_TC_FILTER")) ctx->tc_force_filter = (e[0] == 't') ? 1 : (e[0] == 'p' ? 0 : -1);
     if (const char* e = std::getenv("GMM_TC_FLUSH")) ctx->tc_flush = std::atoi(e);
+    if (const char* e = std::getenv("GMM_WIDE_PIECE")) {
+        const long long v = std::atoll(e);
+        if (v >= 256 && v <= WIDE_PIECE) ctx->wide_piece = v / 256 * 256;
+    }
     if (const char* e = std::getenv("GMM_TC_PIECE")) {
         const long long v = std::atoll(e);
         if (v >= 64 && v <= TC_YPOINTS) ctx->tc_piece = v / 64 * 64;
@@ -767,9 +866,11 @@ int assign_topm_impl(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, cons
 }
 }  // namespace
 
-int gmm_tensor_path_supports(int D, int K) { return tc_supports(D, K) ? 1 : 0; }
+int gmm_tensor_path_supports(int D, int K) { return (tc_supports(D, K) || wide_supports(D, K)) ? 1 : 0; }
 
-int gmm_auto_path(int D, int K) { return auto_is_tensor(D, K) ? GMM_PATH_TENSOR : GMM_PATH_FP32; }
+int gmm_auto_path(int D, int K) {
+    return (auto_is_tensor(D, K) || (wide_supports(D, K) && K >= 64)) ? GMM_PATH_TENSOR : GMM_PATH_FP32;
+}
 
 size_t gmm_scratch_bytes(int D, int K) {
     if (D < 1 || K < 1) return 0;
@@ -961,7 +1062,7 @@ int gmm_fisher_vectors(gmm_ctx* ctx, const float* X, int64_t N, const int64_t* o
     int64_t total_points = 0;
     for (int g = 0; g < G; ++g) total_points += offsets[g + 1] - offsets[g];
     CHECK(prepare_and_choose(ctx, total_points > 0 ? total_points : 1, D, K, pi, mu, var, &path));
-    if (path == GMM_PATH_TENSOR && ctx->path == GMM_PATH_AUTO) {
+    if (path == GMM_PATH_TENSOR && ctx->path == GMM_PATH_AUTO && !wide_supports(D, K)) {
         // Once the limit flags nearly all the components the tile kernel has no well-conditioned logits left to bound
         // a point's maximum with, tests every pair exactly, and the FP32 kernels are the faster exact path.
         int n_ill = 0;
@@ -977,7 +1078,7 @@ int gmm_fisher_vectors(gmm_ctx* ctx, const float* X, int64_t N, const int64_t* o
     // order of size so that the groups of a launch finish together.  Larger groups go one at a time through the step's
     // own accumulation below.
     std::vector<char> batched((size_t)G, 0);
-    if (path == GMM_PATH_TENSOR) {
+    if (path == GMM_PATH_TENSOR && !wide_supports(D, K)) {      // (D > 128: every group goes through the step's own two sweeps below)
         const TcBuffers tb = ctx->tc();
         const TcPlan pl = tc_plan(D, K, 160);
         const int Qmax = ctx->tc_Q;

@@ -525,8 +525,7 @@ def test_data_far_from_the_origin(fg, ctx):
         got = _gpu_step(ctx, _t(X), pi, mu, var)
         what = f"path {path}, data far from the origin"
         assert abs(got[3] - ref[3]) <= 1e-5 * abs(ref[3]), path
-        for g_, r_ in zip(got[:3], ref[:3]):            # raw statistics: 1e-6 of their own size
-            assert np.abs(g_ - r_).max() <= 1e-6 * np.abs(r_).max() + 1e-9, what
+        assert_stats_close(N, s, got[:3], ref[:3], what)
         pi_d, mu_d, var_d = _t(pi), _t(mu), _t(var)
         ctx.gmm_finalize(N, _t(got[0], torch.float64), _t(got[1], torch.float64), _t(got[2], torch.float64), 1e-6,
                          pi_d, mu_d, var_d)

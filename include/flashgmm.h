@@ -78,6 +78,9 @@ int gmm_tensor_path_supports(int D, int K);
 int gmm_auto_path(int D, int K);
 /* The path (GMM_PATH_FP32 or GMM_PATH_TENSOR) the most recent compute call actually ran. */
 int gmm_last_path(const gmm_ctx* ctx);
+/* How many components the most recent tensor-path step treated as ill-conditioned, i.e. evaluated (where they matter)
+ * exactly in fp32 instead of through the expanded quadratic form; 0 after a step on the FP32 path. */
+int gmm_last_exact_count(const gmm_ctx* ctx);
 
 /* E-step and sufficient statistics under the INPUT parameters (paper Section 2 responsibilities; Eq. 1; the
  * numerators of Eq. 2 and Eq. 3; Algorithm 1 without its last line).

@@ -43,11 +43,17 @@ __device__ __forceinline__ float fast_ex2(float x) {
 // ACC = float: one fp32 accumulation chain over D (D <= 128: a few 1e-6 of error).  ACC = double: each 32-dimension
 // chunk is summed in fp32 and the chunk sums are added in float64, which keeps long chains (D = 768: |q| ~ 1000 in the
 // log2 domain) from drowning the responsibilities in rounding noise.
-template <typename ACC>
+// EARLY: cv[b] = constant of this thread's component b, fl[a] = a value below which log2 z of this thread's point a is
+// negligible (a lower bound of the point's log2 Z minus 40).  The quadratic forms only grow with every chunk of
+// dimensions, so once cv - q < fl for every pair of the tile the rest of the chunks cannot matter: the block leaves the
+// loop together and the caller sees q = +inf (log2 z = -inf).  This is what makes a sub-mixture of collapsed components
+// (hopeless for every point but their own) cost one chunk per tile instead of D / 32.
+template <typename ACC, bool EARLY = false>
 __device__ __forceinline__ void tile_quadratic(TileSmem& sm, const float* __restrict__ X, int64_t row0, int64_t n,
                                                int D, const float* __restrict__ mu, const float* __restrict__ w2,
                                                int k0, int K, ACC (&q)[4][4], const float* __restrict__ g,
-                                               const int32_t* __restrict__ gather = nullptr) {
+                                               const int32_t* __restrict__ gather = nullptr, const ACC* cv = nullptr,
+                                               const ACC* fl = nullptr) {
     constexpr bool HP = sizeof(ACC) == 8;
     const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
 #pragma unroll
@@ -136,6 +142,20 @@ __device__ __forceinline__ void tile_quadratic(TileSmem& sm, const float* __rest
         for (int a = 0; a < 4; ++a)
 #pragma unroll
             for (int b = 0; b < 4; ++b) q[a][b] = HP ? (ACC)(q[a][b] + (ACC)part[a][b]) : (ACC)part[a][b];
+        if (EARLY && d0 + DCH < D) {
+            bool live = false;
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+#pragma unroll
+                for (int b = 0; b < 4; ++b) live |= (cv[b] - q[a][b] >= fl[a]);
+            if (!__syncthreads_or(live ? 1 : 0)) {
+#pragma unroll
+                for (int a = 0; a < 4; ++a)
+#pragma unroll
+                    for (int b = 0; b < 4; ++b) q[a][b] = (ACC)CUDART_INF_F;
+                return;
+            }
+        }
     }
 }
 
@@ -171,7 +191,7 @@ __device__ __forceinline__ void lse_tile(unsigned char* smem_raw, int64_t blk, c
                                          const float* __restrict__ mu, const float* __restrict__ w2, const double* __restrict__ c2,
                                          const float* __restrict__ g, double* __restrict__ logZ2, double* __restrict__ llpart,
                                          int m_out, int32_t* __restrict__ idx_out, float* __restrict__ resp_out,
-                                         const int32_t* __restrict__ gather) {
+                                         const int32_t* __restrict__ gather, const double* __restrict__ lower2 = nullptr) {
     TileSmem& sm = *reinterpret_cast<TileSmem*>(smem_raw);
     __shared__ double ll_s[TP];
     const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
@@ -188,15 +208,25 @@ __device__ __forceinline__ void lse_tile(unsigned char* smem_raw, int64_t blk, c
         for (int a = 0; a < 4; ++a) top[a].init();
     }
 
+    // lower2 (only with EARLY instantiations: M == 0, ACC = double): a lower bound of every point's final log2 Z, known
+    // from elsewhere (the other components' log-sum-exp); terms more than 2^-40 below it are not evaluated to the end
+    constexpr bool EARLY = (M == 0) && (sizeof(ACC) == 8);
+    ACC fl[4];
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+        const int64_t row = row0 + 4 * ty + a;
+        fl[a] = (EARLY && lower2) ? ((row < n) ? (ACC)(__ldg(lower2 + row) - 40.0) : (ACC)CUDART_INF_F) : NEG_INF;
+    }
     for (int k0 = 0; k0 < K; k0 += TC) {
         ACC q[4][4];
-        tile_quadratic<ACC>(sm, X, row0, n, D, mu, w2, k0, K, q, g, gather);
         ACC cv[4];
 #pragma unroll
         for (int b = 0; b < 4; ++b) {
             const int k = k0 + 4 * tx + b;
             cv[b] = (k < K) ? (ACC)__ldg(c2 + k) : NEG_INF;
         }
+        if (EARLY && lower2) tile_quadratic<ACC, EARLY>(sm, X, row0, n, D, mu, w2, k0, K, q, g, gather, cv, fl);
+        else tile_quadratic<ACC>(sm, X, row0, n, D, mu, w2, k0, K, q, g, gather);
 #pragma unroll
         for (int a = 0; a < 4; ++a) {
             ACC l[4];
@@ -296,12 +326,12 @@ lse_kernel(const float* __restrict__ X, int64_t n, int D, int K, const float* __
            const float* __restrict__ w2, const double* __restrict__ c2, const float* __restrict__ g,
            double* __restrict__ logZ2, double* __restrict__ llpart, int m_out, int32_t* __restrict__ idx_out,
            float* __restrict__ resp_out, const int* __restrict__ run_if, const int32_t* __restrict__ gather,
-           const int* __restrict__ gather_count) {
+           const int* __restrict__ gather_count, const double* __restrict__ lower2 = nullptr) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     // run_if: the launch does nothing unless run_if[0] != 0 (the tensor-core assignment covers the other case)
     if (run_if && run_if[0] == 0) return;
     if (!gather) {                                   // one CTA per tile
-        lse_tile<M, ACC>(smem_raw, blockIdx.x, X, n, D, K, mu, w2, c2, g, logZ2, llpart, m_out, idx_out, resp_out, nullptr);
+        lse_tile<M, ACC>(smem_raw, blockIdx.x, X, n, D, K, mu, w2, c2, g, logZ2, llpart, m_out, idx_out, resp_out, nullptr, lower2);
         return;
     }
     // gather: the points are X[gather[0 .. *gather_count)] (top-m outputs go to those rows).  The count is only known on
@@ -426,6 +456,9 @@ mstep_kernel(const float* __restrict__ X, int64_t n, int D, int K, const float* 
 constexpr int WT = 3;
 constexpr size_t MSTEP_WIDE_SMEM = sizeof(TileSmem) + (size_t)WT * TP * LDR * 4 + (size_t)TP * LDX * 4;
 
+// EARLY: tiles none of whose (point, component) pairs can reach 2^-40 of the point's Z leave the quadratic form after the
+// first chunks (see tile_quadratic); batches in which every responsibility is zero skip the sweep over D as well.
+template <bool EARLY>
 __global__ void __launch_bounds__(NTHREADS, 2)
 mstep_wide_kernel(const float* __restrict__ X, int64_t n, int D, int K, const float* __restrict__ mu,
                   const float* __restrict__ w2, const double* __restrict__ c2, const float* __restrict__ g,
@@ -456,13 +489,24 @@ mstep_wide_kernel(const float* __restrict__ X, int64_t n, int D, int K, const fl
     for (int64_t t0 = split; t0 < ntiles; t0 += (int64_t)nsplits * WT) {
         // ---- responsibilities of the batch (tiles t0, t0 + nsplits, ...) ----
         int nb = 0;
+        bool any_r = false;
         for (int w = 0; w < WT; ++w) {
             const int64_t t = t0 + (int64_t)w * nsplits;
             if (t >= ntiles) break;
             ++nb;
             const int64_t row0 = t * TP;
             double q[4][4];
-            tile_quadratic<double>(sm, X, row0, n, D, mu, w2, k0, K, q, g);
+            if (EARLY) {
+                double fl[4];
+#pragma unroll
+                for (int a = 0; a < 4; ++a) {
+                    const int64_t row = row0 + 4 * ty + a;
+                    fl[a] = (row < n) ? __ldg(logZ2 + row) - 40.0 : (double)CUDART_INF_F;
+                }
+                tile_quadratic<double, true>(sm, X, row0, n, D, mu, w2, k0, K, q, g, nullptr, cv, fl);
+            } else {
+                tile_quadratic<double>(sm, X, row0, n, D, mu, w2, k0, K, q, g);
+            }
             float* r_s = r_all + w * TP * LDR;
 #pragma unroll
             for (int a = 0; a < 4; ++a) {
@@ -473,10 +517,15 @@ mstep_wide_kernel(const float* __restrict__ X, int64_t n, int D, int K, const fl
                 rv.y = fast_ex2((float)(cv[1] - q[a][1] - lz));
                 rv.z = fast_ex2((float)(cv[2] - q[a][2] - lz));
                 rv.w = fast_ex2((float)(cv[3] - q[a][3] - lz));
+                any_r |= (rv.x > 0.f) || (rv.y > 0.f) || (rv.z > 0.f) || (rv.w > 0.f);
                 *reinterpret_cast<float4*>(&r_s[(4 * ty + a) * LDR + 4 * tx]) = rv;
             }
         }
-        __syncthreads();
+        if (EARLY) {
+            if (!__syncthreads_or(any_r ? 1 : 0)) continue;          // nothing to accumulate from this batch
+        } else {
+            __syncthreads();
+        }
         if (tid < TC) {
             float s = 0.f;
             for (int w = 0; w < nb; ++w)
@@ -659,10 +708,11 @@ cudaError_t launch_prepare_fp32(cudaStream_t s, int D, int K, const float* pi, c
 static inline bool fp32_high_precision(int D) { return D > 128; }
 
 cudaError_t launch_lse_fp32(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu,
-                            const float* w2, const double* c2d, const float* g, double* logZ2, double* llpart) {
+                            const float* w2, const double* c2d, const float* g, double* logZ2, double* llpart,
+                            const double* lower2) {
     const unsigned blocks = (unsigned)((n + TP - 1) / TP);
     if (fp32_high_precision(D))
-        lse_kernel<0, double><<<blocks, NTHREADS, sizeof(TileSmem), s>>>(X, n, D, K, mu, w2, c2d, g, logZ2, llpart, 0, nullptr, nullptr, nullptr, nullptr, nullptr);
+        lse_kernel<0, double><<<blocks, NTHREADS, sizeof(TileSmem), s>>>(X, n, D, K, mu, w2, c2d, g, logZ2, llpart, 0, nullptr, nullptr, nullptr, nullptr, nullptr, lower2);
     else
         lse_kernel<0, float><<<blocks, NTHREADS, sizeof(TileSmem), s>>>(X, n, D, K, mu, w2, c2d, g, logZ2, llpart, 0, nullptr, nullptr, nullptr, nullptr, nullptr);
     return cudaGetLastError();
@@ -711,15 +761,17 @@ cudaError_t launch_topm_fp32(cudaStream_t s, const float* X, int64_t n, int D, i
 
 cudaError_t launch_mstep_fp32(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu,
                               const float* w2, const double* c2d, const float* g, const double* logZ2, float* partials,
-                              const Fp32Plan& plan) {
+                              const Fp32Plan& plan, bool early) {
     if (plan.wide) {
-        cudaError_t e = cudaFuncSetAttribute(mstep_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)MSTEP_WIDE_SMEM);
+        cudaError_t e = early ? cudaFuncSetAttribute(mstep_wide_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)MSTEP_WIDE_SMEM)
+                              : cudaFuncSetAttribute(mstep_wide_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)MSTEP_WIDE_SMEM);
         if (e != cudaSuccess) return e;
         const size_t bytes = (size_t)plan.splits * ((size_t)K + 2 * (size_t)K * D) * sizeof(double);
         e = cudaMemsetAsync(partials, 0, bytes, s);          // the kernel accumulates into its partials
         if (e != cudaSuccess) return e;
         dim3 wgrid(plan.comp_blocks, plan.splits, 1);
-        mstep_wide_kernel<<<wgrid, NTHREADS, MSTEP_WIDE_SMEM, s>>>(X, n, D, K, mu, w2, c2d, g, logZ2, reinterpret_cast<double*>(partials));
+        if (early) mstep_wide_kernel<true><<<wgrid, NTHREADS, MSTEP_WIDE_SMEM, s>>>(X, n, D, K, mu, w2, c2d, g, logZ2, reinterpret_cast<double*>(partials));
+        else mstep_wide_kernel<false><<<wgrid, NTHREADS, MSTEP_WIDE_SMEM, s>>>(X, n, D, K, mu, w2, c2d, g, logZ2, reinterpret_cast<double*>(partials));
         return cudaGetLastError();
     }
     dim3 grid(plan.comp_blocks, plan.splits, plan.d_chunks);

@@ -6,8 +6,10 @@
 // (128 x 2D x 2 fp16 planes) no longer fits shared memory, so neither can stay on chip for the life of a CTA.
 //
 //   sweep 1  (lse_wide_kernel, TMEM lanes = POINTS)   Algorithm 1, Step 1.  A CTA takes tiles of 128 points and walks the
-//            components in groups of 512 (all 512 TMEM columns as accumulators); for every 64-column atom of the
-//            contraction it streams the tile's Y atom and the group's coefficient atoms through a ring in shared memory.
+//            components in groups of 256 (256 TMEM columns for the main product, 256 for the two small cross products:
+//            the same split, and the same order of accumulation, as in sweep 2, so that both sweeps see the same logits
+//            and the responsibilities of a point sum to one); for every 64-column atom of the contraction it streams the
+//            tile's Y atom and the group's coefficient atoms through a ring in shared memory.
 //            A softmax thread owns one point: running (max, sum) over all K, log2 Z_i to a scratch buffer of one piece
 //            (2^17 points; no O(N) memory), sum of log2 Z for the log-likelihood.
 //   sweep 2  (em_wide_kernel, TMEM lanes = COMPONENTS)   Algorithm 1, Step 2.  A CTA owns 128 components and takes
@@ -44,7 +46,7 @@ constexpr float RSCALE = TC_RSCALE;
 
 // ------------------------------------------------------------------------------------------------------------------
 // Sweep 1
-constexpr int L_SLOTS = 7;
+constexpr int L_SLOTS = 6;                          // two steps (Y atom + two coefficient atoms) in flight
 constexpr int L_BAR = L_SLOTS * SLOT;
 constexpr int L_MERGE = L_BAR + 256;                // 128 x 8 bytes: (max, sum) pairs of warpgroup 1, later the log-likelihood terms
 constexpr int L_SMEM = L_MERGE + 1024 + 1024;
@@ -58,6 +60,7 @@ struct LseParams {
     const double* cref;
     double* logz;
     double* llpart;
+    float4* top;         // [n] per point: its two largest approximate log2 z (relative to c_ref) and their components
     int* status;
 };
 
@@ -72,12 +75,13 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
     volatile int* drain_flag = &drain_s;
     float2* merge_s = reinterpret_cast<float2*>(smem + L_MERGE);
     double* ll_s = reinterpret_cast<double*>(smem + L_MERGE);      // after the last tile
+    __shared__ float4 top_s[128];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int64_t ntiles = (p.n + WIDE_TILE - 1) / WIDE_TILE;
     const int64_t ntl = ((int64_t)blockIdx.x < ntiles) ? (ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
     const int NC = p.NC, NZ = p.NZ;
-    const int NG = (NC + 3) >> 2;
+    const int NG = (NC + 1) >> 1;                        // groups of two chunks
 
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L_BAR);
     auto BAR = [&](int i) { return smem_u32(&bars[i]); };
@@ -101,8 +105,8 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
 
     if (warp < 8) {
         // =========================== softmax warps: thread = TMEM lane = point ===========================
-        // Warpgroup g reads chunks 2 g and 2 g + 1 of every group of four chunks; the two running (max, sum) pairs of a
-        // point are merged at the end of its tile.
+        // Warpgroup g reads chunk g of every group of two chunks (main product in columns [128 g, 128 g + 128), cross products
+        // in [256 + 128 g, ...)); the two running (max, sum) pairs of a point are merged at the end of its tile.
         const int grp = warp >> 2, wq = warp & 3;
         const uint32_t lane_addr = ((uint32_t)(wq * 32)) << 16;
         const int pt = wq * 32 + lane;                       // point within the tile
@@ -112,36 +116,47 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
         for (int64_t i = 0; i < ntl; ++i) {
             const int64_t row = (blockIdx.x + i * gridDim.x) * WIDE_TILE + pt;
             float m_run = -1e30f, s_run = 0.f;               // finite start: blocks of -inf logits must not make NaN
+            float t1 = -CUDART_INF_F, t2 = -CUDART_INF_F;    // the two largest logits of this thread's chunks, and where
+            int i1 = -1, i2 = -1;
             for (int g = 0; g < NG; ++g) {
-                const int nch = (NC - 4 * g < 4) ? (NC - 4 * g) : 4;
+                const int nch = (NC - 2 * g < 2) ? (NC - 2 * g) : 2;
                 const bool got = bar_wait(BAR(LB_LFULL), uses & 1u, abort_flag, p.status, false);
                 const bool ok = __all_sync(0xffffffffu, got);
                 fence_after();
                 ++uses;
                 if (ok) {
-#pragma unroll 1
-                    for (int cc = 0; cc < 2; ++cc) {
-                        const int c = 2 * grp + cc;
-                        if (c >= nch) break;                 // uniform over the warpgroup
+                    {
+                        const int c = grp;
+                        if (c < nch) {                       // uniform over the warpgroup
 #pragma unroll 1
                         for (int sub = 0; sub < 4; ++sub) {
-                            uint32_t v[32];
+                            uint32_t v[32], vc[32];
                             tmem_ld32(tmem + c * 128 + sub * 32 + lane_addr, v);
+                            tmem_ld32(tmem + 256 + c * 128 + sub * 32 + lane_addr, vc);
                             tmem_wait_ld();
-                            const int col0 = (4 * g + c) * 128 + sub * 32;
+                            const int col0 = (2 * g + c) * 128 + sub * 32;
                             const float4* tc4 = reinterpret_cast<const float4*>(p.tkck + col0);
                             float l[32];
                             float bmax = -CUDART_INF_F;
 #pragma unroll
                             for (int j = 0; j < 32; j += 2) {
                                 const float4 q = __ldg(tc4 + (j >> 1));          // (t, c) of two components; same address in every lane
-                                l[j] = fmaf(__uint_as_float(v[j]), q.x, q.y);
-                                l[j + 1] = fmaf(__uint_as_float(v[j + 1]), q.z, q.w);
+                                l[j] = fmaf(__uint_as_float(v[j]) + __uint_as_float(vc[j]), q.x, q.y);
+                                l[j + 1] = fmaf(__uint_as_float(v[j + 1]) + __uint_as_float(vc[j + 1]), q.z, q.w);
                                 bmax = fmaxf(bmax, fmaxf(l[j], l[j + 1]));
                             }
                             if (bmax > m_run) {
                                 s_run *= fast_ex2(m_run - bmax);
                                 m_run = bmax;
+                            }
+                            if (bmax > t2) {                 // (rare after the first chunks)
+#pragma unroll
+                                for (int j = 0; j < 32; ++j) {
+                                    if (l[j] > t2) {
+                                        if (l[j] > t1) { t2 = t1; i2 = i1; t1 = l[j]; i1 = col0 + j; }
+                                        else { t2 = l[j]; i2 = col0 + j; }
+                                    }
+                                }
                             }
                             float acc0 = 0.f, acc1 = 0.f;
 #pragma unroll
@@ -151,21 +166,36 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
                             }
                             s_run += acc0 + acc1;
                         }
+                        }
                     }
                 }
                 fence_before();
                 bar_arrive(BAR(LB_LEMPTY));
             }
-            // merge the two warpgroups' pairs; warpgroup 0 writes log2 Z
-            if (grp == 1) merge_s[pt] = make_float2(m_run, s_run);
+            // merge the two warpgroups' pairs; warpgroup 0 writes log2 Z and the two leading candidates
+            if (grp == 1) {
+                merge_s[pt] = make_float2(m_run, s_run);
+                top_s[pt] = make_float4(t1, t2, __int_as_float(i1), __int_as_float(i2));
+            }
             named_bar_sync(1, 256);
             if (grp == 0) {
                 const float2 o = merge_s[pt];
                 const float m = fmaxf(m_run, o.x);
                 const float s = s_run * fast_ex2(m_run - m) + o.y * fast_ex2(o.x - m);
+                const float4 ot = top_s[pt];
+                const float ov[2] = {ot.x, ot.y};
+                const int oi[2] = {__float_as_int(ot.z), __float_as_int(ot.w)};
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                    if (ov[j] > t2) {
+                        if (ov[j] > t1) { t2 = t1; i2 = i1; t1 = ov[j]; i1 = oi[j]; }
+                        else { t2 = ov[j]; i2 = oi[j]; }
+                    }
+                }
                 if (row < p.n && !*abort_flag) {
                     const double lz = cref + (double)m + (double)log2f(s);
                     p.logz[row] = lz;
+                    p.top[row] = make_float4(t1, t2, __int_as_float(i1), __int_as_float(i2));
                     ll_acc += lz;
                 }
             }
@@ -173,7 +203,7 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
         }
         if (grp == 0) ll_s[pt] = ll_acc;
         named_bar_sync(1, 256);
-        if (tid == 0) {
+        if (tid == 0 && p.llpart) {
             double s = 0.0;
             for (int j = 0; j < 128; ++j) s += ll_s[j];
             p.llpart[blockIdx.x] += s * 0.69314718055994530942;       // one owner per slot: launches add up
@@ -204,10 +234,10 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
         for (int64_t i = 0; i < ntl && ok; ++i) {
             const int32_t row0 = (int32_t)((blockIdx.x + i * gridDim.x) * WIDE_TILE);
             for (int gq = 0; gq < NG && ok; ++gq) {
-                const int nch = (NC - 4 * gq < 4) ? (NC - 4 * gq) : 4;
+                const int nch = (NC - 2 * gq < 2) ? (NC - 2 * gq) : 2;
                 for (int z = 0; z < NZ && ok; ++z) {
                     ok = item(&tm_yhi, &tm_ylo, row0, z);
-                    for (int c = 0; c < nch && ok; ++c) ok = item(&tm_phi, &tm_plo, (4 * gq + c) * 128, z);
+                    for (int c = 0; c < nch && ok; ++c) ok = item(&tm_phi, &tm_plo, (2 * gq + c) * 128, z);
                 }
             }
         }
@@ -234,7 +264,7 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
         uint32_t groups_done = 0;
         for (int64_t i = 0; i < ntl && alive; ++i) {
             for (int gq = 0; gq < NG && alive; ++gq) {
-                const int nch = (NC - 4 * gq < 4) ? (NC - 4 * gq) : 4;
+                const int nch = (NC - 2 * gq < 2) ? (NC - 2 * gq) : 2;
                 if (groups_done > 0 && !wait_all(BAR(LB_LEMPTY), (groups_done - 1) & 1u)) { alive = false; break; }
                 for (int z = 0; z < NZ && alive; ++z) {
                     const int sy = (int)(g % L_SLOTS);
@@ -247,14 +277,15 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
                         if (elect_one()) {
                             const uint64_t ah = d0 + ((sy * SLOT) >> 4), al = ah + ((SLOT / 2) >> 4);
                             const uint64_t bh = d0 + ((sp * SLOT) >> 4), bl = bh + ((SLOT / 2) >> 4);
-                            const uint32_t d = tmem + c * 128;
-                            // the two small cross products of the atom first, then the leading one
+                            const uint32_t d = tmem + c * 128, dc = tmem + 256 + c * 128;
+                            // the two small cross products into their own accumulator, the leading product into the main one:
+                            // the same three chains, in the same order, as the E-step of sweep 2
 #pragma unroll
-                            for (int j = 0; j < 4; ++j) mma_ss(d, ah + ((j * 32) >> 4), bl + ((j * 32) >> 4), idesc, (z > 0 || j > 0) ? 1u : 0u);
+                            for (int j = 0; j < 4; ++j) mma_ss(dc, ah + ((j * 32) >> 4), bl + ((j * 32) >> 4), idesc, (z > 0 || j > 0) ? 1u : 0u);
 #pragma unroll
-                            for (int j = 0; j < 4; ++j) mma_ss(d, al + ((j * 32) >> 4), bh + ((j * 32) >> 4), idesc, 1u);
+                            for (int j = 0; j < 4; ++j) mma_ss(dc, al + ((j * 32) >> 4), bh + ((j * 32) >> 4), idesc, 1u);
 #pragma unroll
-                            for (int j = 0; j < 4; ++j) mma_ss(d, ah + ((j * 32) >> 4), bh + ((j * 32) >> 4), idesc, 1u);
+                            for (int j = 0; j < 4; ++j) mma_ss(d, ah + ((j * 32) >> 4), bh + ((j * 32) >> 4), idesc, (z > 0 || j > 0) ? 1u : 0u);
                             mma_commit(BAR(LB_EMPTY + sp));
                             if (c == nch - 1) mma_commit(BAR(LB_EMPTY + sy));
                             if (c == nch - 1 && z == NZ - 1) mma_commit(BAR(LB_LFULL));
@@ -284,8 +315,8 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
 // Sweep 2
 constexpr int E_SLOTS = 6;
 constexpr int E_BAR = E_SLOTS * SLOT;
-constexpr int E_LZ = E_BAR + 256;                  // 2 x 256 floats: log2 Z - c_ref of the batch's points
-constexpr int E_SMEM = E_LZ + 2048 + 1024;
+constexpr int E_LZ = E_BAR + 256;                  // 2 x 256 doubles: log2 Z of the batch's points
+constexpr int E_SMEM = E_LZ + 4096 + 1024;
 enum { EB_FULL = 0, EB_EMPTY = E_SLOTS, EB_LFULL = 2 * E_SLOTS, EB_RREADY, EB_ACCFULL0, EB_ACCFULL1, EB_ACCFREE0,
        EB_ACCFREE1, EB_FINAL, EB_COUNT };
 
@@ -293,7 +324,7 @@ struct EmWideParams {
     int64_t n;
     int CL, R, NZ, pcols;
     const float2* tkck;
-    const double* cref;
+    const double* ckd;
     const double* logz;
     float* partial;      // [R * CL][pcols][128]
     int* status;
@@ -349,16 +380,17 @@ em_wide_kernel(const EmWideParams p, const __grid_constant__ CUtensorMap tm_phi,
         const uint32_t lane_addr = ((uint32_t)(wq * 32)) << 16;
         const int kloc = wq * 32 + lane;
         const float2 tc = __ldg(p.tkck + slice * 128 + kloc);
-        const double cref = *p.cref;
-        float* lz_s = reinterpret_cast<float*>(smem + E_LZ);              // [2][256]
+        // c_k - log2 Z_i is formed in float64 (both are in the thousands, their difference is what the exponent needs)
+        const double ckd = (tc.y == -CUDART_INF_F) ? -CUDART_INF : __ldg(p.ckd + slice * 128 + kloc);
+        double* lz_s = reinterpret_cast<double*>(smem + E_LZ);            // [2][256]
         float* pblk = p.partial + (size_t)blockIdx.x * p.pcols * 128 + kloc;      // [column][component]: one owner per address
         uint32_t acc_uses[2] = {0u, 0u};
         for (int64_t b = 0; b < nbl; ++b) {
             const int64_t row0 = (range + b * p.R) * WIDE_BATCH;
-            float* lz = lz_s + (b & 1) * 256;
-            {   // log2 Z - c_ref of the batch's points (+inf beyond n: those points get r = 0)
+            double* lz = lz_s + (b & 1) * 256;
+            {   // log2 Z of the batch's points (+inf beyond n: those points get r = 0)
                 const int64_t row = row0 + (tid & 255);
-                lz[tid & 255] = (row < p.n) ? (float)(p.logz[row] - cref) : CUDART_INF_F;
+                lz[tid & 255] = (row < p.n) ? p.logz[row] : CUDART_INF;
             }
             named_bar_sync(1, 256);
             const bool got = bar_wait(BAR(EB_LFULL), (uint32_t)(b & 1), abort_flag, p.status, false);
@@ -376,13 +408,14 @@ em_wide_kernel(const EmWideParams p, const __grid_constant__ CUtensorMap tm_phi,
                     uint32_t hi[16], lo[16];
 #pragma unroll
                     for (int j = 0; j < 32; j += 4) {
-                        const float4 z4 = *reinterpret_cast<const float4*>(lz + p0 + j);
+                        const double2 za = *reinterpret_cast<const double2*>(lz + p0 + j);
+                        const double2 zb = *reinterpret_cast<const double2*>(lz + p0 + j + 2);
                         float r[4];
-                        const float zz[4] = {z4.x, z4.y, z4.z, z4.w};
+                        const double zz[4] = {za.x, za.y, zb.x, zb.y};
 #pragma unroll
                         for (int q = 0; q < 4; ++q) {
                             const float acc = __uint_as_float(vm[j + q]) + __uint_as_float(vc[j + q]);
-                            r[q] = fast_ex2(fmaf(acc, tc.x, tc.y - zz[q])) * RSCALE;
+                            r[q] = fast_ex2(fmaf(acc, tc.x, (float)(ckd - zz[q]))) * RSCALE;
                         }
                         const __half2 h01 = __floats2half2_rn(r[0], r[1]), h23 = __floats2half2_rn(r[2], r[3]);
                         const float2 b01 = __half22float2(h01), b23 = __half22float2(h23);
@@ -723,7 +756,7 @@ __global__ void __launch_bounds__(256) wide_prepare_kernel(int D, int Dpad, int 
                                                            const float* __restrict__ gd, __half* __restrict__ p_hi,
                                                            __half* __restrict__ p_lo, float* __restrict__ tk,
                                                            double* __restrict__ ckd, float* __restrict__ illb,
-                                                           float cond_limit, int* __restrict__ flags) {
+                                                           float cond_limit, float min_weight, int* __restrict__ flags) {
     extern __shared__ double ab_s[];                     // [2][Dpad]: a, b of this component
     __shared__ double red[4][256];
     const int k = blockIdx.x, t = threadIdx.x;
@@ -783,9 +816,13 @@ __global__ void __launch_bounds__(256) wide_prepare_kernel(int D, int Dpad, int 
         }
         // error estimate of the approximate log2 z: operand rounding at 2^-22 of every term, terms of independent sign
         const double est = 4.0 * 2.384185791015625e-07 * sqrt(red[2][0]);
+        // A component that holds few points (pi_k N below a threshold) is evaluated exactly as well: its parameters are
+        // averages over few responsibilities, which for a component far from most of its points are formed from large
+        // accumulators (|log2 z - c_k| in the thousands) whose truncation error nothing averages out.
         float margin = 0.f;
-        if (k < K && !(est <= (double)cond_limit)) {
-            margin = (float)fmin(8.0 * est, 1e30);
+        if (k < K && pi[k] > 0.f && (!(est <= (double)cond_limit) || pi[k] < min_weight)) {
+            // (flagged for its weight alone: a tiny positive mark, which the list kernel uses to keep the two kinds apart)
+            margin = !(est <= (double)cond_limit) ? (float)fmin(fmax(8.0 * est, 1e-10), 1e30) : 1e-30f;
             if (!(margin > 0.f)) margin = 1e30f;
             atomicOr(flags, 1);
             atomicAdd(flags + 4, 1);
@@ -854,6 +891,158 @@ __global__ void wide_reduce_kernel(int D, int K, int CL, int R, int pcols, const
     }
 }
 
+// Exact log2 Z.  The approximate logits carry an error of up to about 1e-3 (the tensor core truncates its fp32 accumulator
+// at every step; the loss grows with the accumulator's magnitude), most of it common to the components that matter for
+// a point, and log2 Z_i from sweep 1 carries the same error: in r = 2^(log2 z - log2 Z) of sweep 2 it cancels, which is why
+// sweep 2 must use the log2 Z of sweep 1 as it is.  The components evaluated EXACTLY (the sub-mixture of the FP32
+// kernels) need an exact normaliser instead, and so does the log-likelihood: the two leading terms of every point are
+// recomputed exactly (fp32 direct differences, chunk sums added in float64: the arithmetic of the FP32 kernels) and a
+// second array gets Z' = Z + sum_c (2^exact_c - 2^approx_c).  One warp per point.
+__global__ void __launch_bounds__(256) wide_refine_kernel(const float* __restrict__ X, int64_t n, int D, int K,
+                                                          const float* __restrict__ mu, const float* __restrict__ w2,
+                                                          const double* __restrict__ c2d, const double* __restrict__ cref,
+                                                          const float4* __restrict__ top, const double* __restrict__ logz,
+                                                          double* __restrict__ logz_x) {
+    const int64_t i = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (i >= n) return;
+    const float4 t = top[i];
+    const double lz = logz[i], cr = *cref;
+    const float av[2] = {t.x, t.y};
+    const int ak[2] = {__float_as_int(t.z), __float_as_int(t.w)};
+    const float* xr = X + i * D;
+    double corr = 0.0;
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+        const int k = ak[c];
+        if (k < 0 || k >= K) continue;                       // warp-uniform
+        const float* mr = mu + (size_t)k * D;
+        const float* wr = w2 + (size_t)k * D;
+        double q = 0.0;
+        for (int d0 = 0; d0 < D; d0 += 128) {                // a lane sums 4 dimensions of each 128 in fp32
+            float part = 0.f;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int d = d0 + lane + 32 * j;
+                if (d < D) {
+                    const float diff = __ldg(xr + d) - __ldg(mr + d);
+                    part = fmaf(diff * diff, __ldg(wr + d), part);
+                }
+            }
+            q += (double)part;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
+        const double exact = __ldg(c2d + k) - q, approx = cr + (double)av[c];
+        corr += exp2(exact - lz) - exp2(approx - lz);
+    }
+    if (lane == 0) {
+        const double f = 1.0 + corr;
+        logz_x[i] = lz + log2(f > 1e-6 ? f : 1e-6);
+    }
+}
+
+// ---- ill-conditioned components: evaluated exactly by the FP32 kernels as a sub-mixture -------------------------------
+// List of the flagged components (illb > 0), at most WIDE_MAX_ILL; one block of 1024 threads.  First, in ascending order,
+// those flagged by their error estimate (mostly components collapsed onto a point: hopeless for every other point, which
+// the FP32 tile routine notices after its first chunk of dimensions -- but only if ALL 64 components of its tile are of
+// that kind), then those flagged for their small weight alone (broad: they need the full evaluation).
+__global__ void __launch_bounds__(1024) wide_ill_list_kernel(int Kpad, const float* __restrict__ illb, int* __restrict__ list,
+                                                             int* __restrict__ flags) {
+    __shared__ int wcount[32];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    int done = 0;
+    for (int kind = 0; kind < 2; ++kind) {
+        for (int base = 0; base < Kpad; base += 1024) {
+            const int k = base + threadIdx.x;
+            const float e = k < Kpad ? illb[k] : 0.f;
+            const bool is = kind == 0 ? (e > 1e-20f) : (e > 0.f && e <= 1e-20f);
+            const unsigned b = __ballot_sync(0xffffffffu, is);
+            __syncthreads();
+            if (lane == 0) wcount[w] = __popc(b);
+            __syncthreads();
+            int before = 0, total = 0;
+            for (int j = 0; j < 32; ++j) {
+                if (j < w) before += wcount[j];
+                total += wcount[j];
+            }
+            const int pos = done + before + __popc(b & ((1u << lane) - 1u));
+            if (is && pos < WIDE_MAX_ILL) list[pos] = k;
+            done += total;
+        }
+        if (kind == 0) {
+            // pad the first kind to a whole tile of 64 components with repeats of... nothing: the second kind simply starts
+            // at the next multiple of 64 (the gap is filled with component -1 = an empty slot)
+            const int padded = (done + 63) & ~63;
+            for (int j = done + threadIdx.x; j < padded && j < WIDE_MAX_ILL; j += 1024) list[j] = -1;
+            done = padded < WIDE_MAX_ILL ? padded : done;
+            if (threadIdx.x == 0) flags[5] = done;            // where the second kind starts
+            __syncthreads();
+        }
+    }
+    if (threadIdx.x == 0) flags[2] = done < WIDE_MAX_ILL ? done : WIDE_MAX_ILL;
+}
+
+// The listed components' rows of mu, w2 and their constants, packed: the sub-mixture the FP32 kernels evaluate.
+__global__ void wide_ill_gather_kernel(int D, int n_ill, const int* __restrict__ list, const float* __restrict__ mu,
+                                       const float* __restrict__ w2, const double* __restrict__ c2d, float* __restrict__ mu_c,
+                                       float* __restrict__ w2_c, double* __restrict__ c2d_c) {
+    const int j = blockIdx.x;
+    if (j >= n_ill) return;
+    const int k = list[j];
+    for (int d = threadIdx.x; d < D; d += blockDim.x) {
+        mu_c[(size_t)j * D + d] = k >= 0 ? mu[(size_t)k * D + d] : 0.f;
+        w2_c[(size_t)j * D + d] = k >= 0 ? w2[(size_t)k * D + d] : 0.f;
+    }
+    if (threadIdx.x == 0) c2d_c[j] = k >= 0 ? c2d[k] : -CUDART_INF;       // an empty slot: log2 z = -inf for every point
+}
+
+// Both log2 Z arrays (the one consistent with the tensor passes' logits, the exact one) take in the sub-mixture's
+// log-sum-exp b: log2(2^a + 2^b) (b may be NULL); per-block sums of the exact log Z (natural log) for the
+// log-likelihood: fixed grid, fixed order inside a block -> deterministic.
+__global__ void __launch_bounds__(256) wide_merge_ll_kernel(int64_t n, double* __restrict__ logz, double* __restrict__ logz_x,
+                                                            const double* __restrict__ logz_ill, double* __restrict__ llpart) {
+    __shared__ double red[256];
+    const int64_t per = (n + gridDim.x - 1) / gridDim.x;
+    const int64_t lo = (int64_t)blockIdx.x * per, hi = (lo + per < n) ? (lo + per) : n;
+    double s = 0.0;
+    for (int64_t i = lo + threadIdx.x; i < hi; i += 256) {
+        double a = logz[i], x = logz_x[i];
+        if (logz_ill) {
+            const double b = logz_ill[i];
+            double m = fmax(a, b);
+            if (m > -CUDART_INF) a = m + log2(exp2(a - m) + exp2(b - m));
+            m = fmax(x, b);
+            if (m > -CUDART_INF) x = m + log2(exp2(x - m) + exp2(b - m));
+            logz[i] = a;
+            logz_x[i] = x;
+        }
+        s += x;
+    }
+    red[threadIdx.x] = s;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) {
+        if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) llpart[blockIdx.x] += red[0] * 0.69314718055994530942;
+}
+
+// The sub-mixture's statistics go to the rows of its components (which the tensor passes left at zero).
+__global__ void wide_ill_scatter_kernel(int D, int K, int n_ill, const int* __restrict__ list, const double* __restrict__ Nk_c,
+                                        const double* __restrict__ S1_c, const double* __restrict__ S2_c, double* __restrict__ Nk,
+                                        double* __restrict__ S1, double* __restrict__ S2) {
+    const int j = blockIdx.x;
+    if (j >= n_ill) return;
+    const int k = list[j];
+    if (k < 0) return;
+    if (threadIdx.x == 0) Nk[k] += Nk_c[j];
+    for (int d = threadIdx.x; d < D; d += blockDim.x) {
+        S1[(size_t)k * D + d] += S1_c[(size_t)j * D + d];
+        S2[(size_t)k * D + d] += S2_c[(size_t)j * D + d];
+    }
+}
+
 // A plane [rows][pitch bytes] seen as a 3-D tensor (x = 64 halves of an atom's row, y = row, z = atom): a box of
 // (64, box_rows, box_atoms) lands in shared memory as [atom][row][128 bytes], each 128-byte row swizzled.
 cudaError_t wide_make_map(CUtensorMap* tm, void* base, int64_t rows, int64_t pitch, int atoms, int box_rows, int box_atoms) {
@@ -898,7 +1087,7 @@ WidePlan wide_plan(int D, int K, int num_sms) {
 }
 
 cudaError_t launch_prepare_wide(cudaStream_t s, int D, int K, const float* pi, const float* mu, const float* var,
-                                const WideBuffers& wb, float cond_limit) {
+                                const WideBuffers& wb, float cond_limit, float min_weight) {
     const WidePlan pl = wide_plan(D, K, 148);
     cudaError_t e = cudaMemsetAsync(wb.flags, 0, 8 * sizeof(int), s);
     if (e != cudaSuccess) return e;
@@ -907,10 +1096,41 @@ cudaError_t launch_prepare_wide(cudaStream_t s, int D, int K, const float* pi, c
     if (e != cudaSuccess) return e;
     wide_prepare_kernel<<<pl.Kpad, 256, (size_t)2 * pl.Dpad * sizeof(double), s>>>(
         D, pl.Dpad, K, pi, mu, var, wb.sd, wb.kap, wb.gd, reinterpret_cast<__half*>(wb.p_hi), reinterpret_cast<__half*>(wb.p_lo),
-        wb.tk, wb.ckd, wb.illb, cond_limit, wb.flags);
+        wb.tk, wb.ckd, wb.illb, cond_limit, min_weight, wb.flags);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     wide_cref_kernel<<<1, 1024, 0, s>>>(pl.Kpad, wb.tk, wb.ckd, wb.illb, wb.cref, reinterpret_cast<float2*>(wb.tkck));
+    return cudaGetLastError();
+}
+
+cudaError_t launch_ill_list_wide(cudaStream_t s, int D, int K, const WideBuffers& wb) {
+    const WidePlan pl = wide_plan(D, K, 148);
+    wide_ill_list_kernel<<<1, 1024, 0, s>>>(pl.Kpad, wb.illb, wb.ill_list, wb.flags);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_ill_gather_wide(cudaStream_t s, int D, int n_ill, const WideBuffers& wb, const float* mu, const float* w2,
+                                   const double* c2d) {
+    wide_ill_gather_kernel<<<(unsigned)n_ill, 256, 0, s>>>(D, n_ill, wb.ill_list, mu, w2, c2d, wb.mu_c, wb.w2_c, wb.c2d_c);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_refine_wide(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu, const float* w2,
+                               const double* c2d, const WideBuffers& wb) {
+    wide_refine_kernel<<<(unsigned)((n + 7) / 8), 256, 0, s>>>(X, n, D, K, mu, w2, c2d, wb.cref, reinterpret_cast<const float4*>(wb.top), wb.logz, wb.logz_x);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_merge_ll_wide(cudaStream_t s, int64_t n, const WideBuffers& wb, const double* logz_ill) {
+    wide_merge_ll_kernel<<<WIDE_LL_BLOCKS, 256, 0, s>>>(n, wb.logz, wb.logz_x, logz_ill, wb.llpart);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_ill_scatter_wide(cudaStream_t s, int D, int K, int n_ill, const WideBuffers& wb, double* Nk, double* S1,
+                                    double* S2) {
+    const size_t KD = (size_t)n_ill * D;
+    wide_ill_scatter_kernel<<<(unsigned)n_ill, 256, 0, s>>>(D, K, n_ill, wb.ill_list, wb.stats_c, wb.stats_c + n_ill,
+                                                            wb.stats_c + n_ill + KD, Nk, S1, S2);
     return cudaGetLastError();
 }
 
@@ -940,7 +1160,8 @@ cudaError_t launch_lse_wide(cudaStream_t s, int64_t n, int D, int K, const WideB
     if (e != cudaSuccess) return e;
     LseParams p;
     p.n = n; p.NC = pl.CL; p.NZ = atoms;
-    p.tkck = reinterpret_cast<const float2*>(wb.tkck); p.cref = wb.cref; p.logz = wb.logz; p.llpart = wb.llpart; p.status = status;
+    p.tkck = reinterpret_cast<const float2*>(wb.tkck); p.cref = wb.cref; p.logz = wb.logz; p.llpart = nullptr; p.status = status;
+    p.top = reinterpret_cast<float4*>(wb.top);
     const int64_t ntiles = (n + WIDE_TILE - 1) / WIDE_TILE;
     const unsigned grid = (unsigned)(ntiles < num_sms ? ntiles : num_sms);
     lse_wide_kernel<<<grid, WT_THREADS, L_SMEM, s>>>(p, tm_yhi, tm_ylo, tm_phi, tm_plo);
@@ -964,7 +1185,7 @@ cudaError_t launch_em_wide(cudaStream_t s, int64_t n, int D, int K, const WideBu
     if (e != cudaSuccess) return e;
     EmWideParams p;
     p.n = n; p.CL = pl.CL; p.R = pl.R; p.NZ = atoms; p.pcols = pl.pcols;
-    p.tkck = reinterpret_cast<const float2*>(wb.tkck); p.cref = wb.cref; p.logz = wb.logz; p.partial = wb.partial; p.status = status;
+    p.tkck = reinterpret_cast<const float2*>(wb.tkck); p.ckd = wb.ckd; p.logz = wb.logz; p.partial = wb.partial; p.status = status;
     em_wide_kernel<<<(unsigned)(pl.CL * pl.R), WT_THREADS, E_SMEM, s>>>(p, tm_phi, tm_plo, tm_ye_hi, tm_ye_lo, tm_ym_hi, tm_ym_lo);
     return cudaGetLastError();
 }

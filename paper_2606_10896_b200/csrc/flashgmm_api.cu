@@ -34,7 +34,7 @@ struct ScratchLayout {
     size_t tc_phi, tc_plo, tc_tk, tc_ck, tc_sd, tc_kap, tc_gd, tc_illb, tc_flags, tc_xg, tc_xl, tc_partial, tc_llpart, tc_partial_bytes, tc_yhi, tc_ylo, tc_phirm, tc_plorm, tc_tkck, tc_illlist, tc_illcache, tc_decdim, tc_decw, tc_decmu;
     bool tc;
     // the tensor-core path for D > 128
-    size_t w_sd, w_kap, w_gd, w_phi, w_plo, w_tk, w_tkck, w_ckd, w_cref, w_illb, w_flags, w_yhi, w_ylo, w_logz, w_partial, w_llpart;
+    size_t w_sd, w_kap, w_gd, w_phi, w_plo, w_tk, w_tkck, w_ckd, w_cref, w_illb, w_flags, w_yhi, w_ylo, w_logz, w_partial, w_llpart, w_illlist, w_muc, w_w2c, w_c2dc, w_statsc, w_top, w_logzx;
     size_t w_partial_bytes;
     bool wide;
 };
@@ -88,7 +88,7 @@ ScratchLayout scratch_layout(int D, int K, bool planes) {
         L.tc_yhi = take(TC_YPLANE_BYTES);
         L.tc_ylo = take(TC_YPLANE_BYTES);
     }
-    L.w_sd = L.w_kap = L.w_gd = L.w_phi = L.w_plo = L.w_tk = L.w_tkck = L.w_ckd = L.w_cref = L.w_illb = L.w_flags = L.w_yhi = L.w_ylo = L.w_logz = L.w_partial = L.w_llpart = 0;
+    L.w_sd = L.w_kap = L.w_gd = L.w_phi = L.w_plo = L.w_tk = L.w_tkck = L.w_ckd = L.w_cref = L.w_illb = L.w_flags = L.w_yhi = L.w_ylo = L.w_logz = L.w_partial = L.w_llpart = L.w_illlist = L.w_muc = L.w_w2c = L.w_c2dc = L.w_statsc = L.w_top = L.w_logzx = 0;
     L.w_partial_bytes = 0;
     L.wide = wide_supports(D, K) && planes;
     if (L.wide) {
@@ -105,9 +105,16 @@ ScratchLayout scratch_layout(int D, int K, bool planes) {
         L.w_illb = take((size_t)wp.Kpad * 4);
         L.w_flags = take(32);
         L.w_logz = take((size_t)WIDE_PIECE * 8);
+        L.w_top = take((size_t)WIDE_PIECE * 16);
+        L.w_logzx = take((size_t)WIDE_PIECE * 8);
         L.w_partial_bytes = (size_t)wp.R * wp.CL * wp.pcols * 128 * 4;
         L.w_partial = take(L.w_partial_bytes);
         L.w_llpart = take(256 * 8);
+        L.w_illlist = take((size_t)WIDE_MAX_ILL * 4);
+        L.w_muc = take((size_t)WIDE_MAX_ILL * D * 4);
+        L.w_w2c = take((size_t)WIDE_MAX_ILL * D * 4);
+        L.w_c2dc = take((size_t)WIDE_MAX_ILL * 8);
+        L.w_statsc = take(((size_t)WIDE_MAX_ILL + 2 * (size_t)WIDE_MAX_ILL * D) * 8);
         L.w_yhi = take((size_t)WIDE_PIECE * wp.Dpad * 4);
         L.w_ylo = take((size_t)WIDE_PIECE * wp.Dpad * 4);
     }
@@ -146,6 +153,11 @@ struct gmm_ctx {
     int64_t tc_piece = TC_YPOINTS;   // points per launch of the tile kernel (<= capacity of the Y planes)
     int64_t wide_piece = WIDE_PIECE; // points per pair of sweeps of the D > 128 tensor path
     int sms = 148;                   // multiprocessors of the device
+    double wide_min_points = 64.0;   // components expected to hold fewer points (pi_k N) are evaluated exactly
+    bool wide_refine = true;         // correct log2 Z by the exact values of each point's two leading terms
+    int wide_n_first = 0;            // of which the first kind (flagged by the error estimate: mostly collapsed components)
+    int wide_n_list = 0;             // slots of the packed sub-mixture (the ill-conditioned components plus padding)
+    int wide_n_ill = 0;              // ill-conditioned components of the current step on the D > 128 tensor path
     int tc_n_ill = 0;                // ill-conditioned components at the last result that was read back (picks the filter)
     int tc_force_filter = -1;        // GMM_TC_FILTER=plain / tight: 0 / 1 (tests); -1: automatic
     int sticky_status = 0;           // status bits read off the device but not yet reported (see ensure_scratch)
@@ -217,8 +229,15 @@ struct gmm_ctx {
         b.y_hi = scratch + lay.w_yhi;
         b.y_lo = scratch + lay.w_ylo;
         b.logz = reinterpret_cast<double*>(scratch + lay.w_logz);
+        b.top = reinterpret_cast<float*>(scratch + lay.w_top);
+        b.logz_x = reinterpret_cast<double*>(scratch + lay.w_logzx);
         b.partial = reinterpret_cast<float*>(scratch + lay.w_partial);
         b.llpart = reinterpret_cast<double*>(scratch + lay.w_llpart);
+        b.ill_list = reinterpret_cast<int*>(scratch + lay.w_illlist);
+        b.mu_c = reinterpret_cast<float*>(scratch + lay.w_muc);
+        b.w2_c = reinterpret_cast<float*>(scratch + lay.w_w2c);
+        b.c2d_c = reinterpret_cast<double*>(scratch + lay.w_c2dc);
+        b.stats_c = reinterpret_cast<double*>(scratch + lay.w_statsc);
         return b;
     }
 };
@@ -369,12 +388,28 @@ int prepare_and_choose(gmm_ctx* ctx, int64_t N, int D, int K, const float* pi, c
         float limit = ctx->tc_cond_limit;
         if (limit < 0.f) limit = ctx->tc_cond_scale * std::sqrt((float)((double)N / (double)K));
         const WideBuffers wb = ctx->wide();
-        KL(launch_prepare_wide(ctx->stream, D, K, pi, mu, var, wb, limit));
+        KL(launch_prepare_wide(ctx->stream, D, K, pi, mu, var, wb, limit, (float)((double)ctx->wide_min_points / (double)N)));
         ctx->launches += 2;
         int n_ill = 0;
         CU(cudaMemcpyAsync(&n_ill, wb.flags + 4, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
         CU(cudaStreamSynchronize(ctx->stream));
-        if (n_ill == 0) *path = GMM_PATH_TENSOR;
+        ctx->wide_n_ill = n_ill;
+        if (n_ill + 64 > WIDE_MAX_ILL || 2 * n_ill > K) return GMM_OK;     // too many: the FP32 kernels take the whole step
+        if (n_ill > 0) {
+            // The flagged components take no part in the tensor passes; the FP32 kernels evaluate them exactly as a packed
+            // sub-mixture (a collapsed component is hopeless for every point but its own, which those kernels notice after
+            // the first 32 dimensions of a tile).
+            KL(launch_ill_list_wide(ctx->stream, D, K, wb));
+            // (the list has a gap of empty slots between its two kinds of components: its length comes back with it)
+            int fl[8];
+            CU(cudaMemcpyAsync(fl, wb.flags, sizeof(fl), cudaMemcpyDeviceToHost, ctx->stream));
+            CU(cudaStreamSynchronize(ctx->stream));
+            const int n_list = fl[2];
+            ctx->wide_n_list = n_list;
+            ctx->wide_n_first = fl[5] < n_list ? fl[5] : n_list;
+            KL(launch_ill_gather_wide(ctx->stream, D, n_list, wb, mu, ctx->w2(), ctx->c2d()));
+        }
+        *path = GMM_PATH_TENSOR;
         return GMM_OK;
     }
     const bool tc_ok = ctx->lay.tc && ctx->tc_Q >= 1;
@@ -410,19 +445,55 @@ int accumulate_points(gmm_ctx* ctx, int path, const float* X, int64_t n, int D, 
         // log-sum-exp, responsibilities + statistics into per-CTA fp32 partials, which are folded into the float64
         // statistics piece by piece (no fp32 chain longer than a piece's batches).
         const WideBuffers wb = ctx->wide();
-        const int grid1 = ctx->sms;
+        const int n_ill = ctx->wide_n_ill > 0 ? ctx->wide_n_list : 0;      // slots of the packed sub-mixture
+        // The sub-mixture's M-step runs as two launches, one per kind of component: tiles of collapsed components leave after
+        // their first chunk of dimensions, so a grid shared with the broad ones would leave most of its CTAs idle.  Each
+        // launch has its own plan; their float64 partials share the FP32 path's partial buffer (sized for all K components).
+        const int n_a = n_ill > 0 ? ctx->wide_n_first : 0, n_b = n_ill - n_a;
+        Fp32Plan plan_a = fp32_plan(D, n_a > 0 ? n_a : 1), plan_b = fp32_plan(D, n_b > 0 ? n_b : 1);
+        if (n_ill > 0) {
+            const size_t cap = fp32_partial_floats(D, K) * sizeof(float);
+            auto fit = [&](Fp32Plan& pl, int kk) {
+                const size_t per_split = ((size_t)kk + 2 * (size_t)kk * D) * sizeof(double);
+                while (pl.splits > 1 && (size_t)pl.splits * per_split > cap) --pl.splits;
+            };
+            if (n_a > 0) fit(plan_a, n_a);
+            if (n_b > 0) fit(plan_b, n_b);
+            CU(cudaMemsetAsync(wb.stats_c, 0, ((size_t)n_ill + 2 * (size_t)n_ill * D) * sizeof(double), ctx->stream));
+        }
         CU(cudaMemsetAsync(wb.llpart, 0, 256 * 8, ctx->stream));
         for (int64_t off = 0; off < n; off += ctx->wide_piece) {
             const int64_t cnt = (n - off < ctx->wide_piece) ? (n - off) : ctx->wide_piece;
+            const float* Xs = X + off * D;
             CU(cudaMemsetAsync(wb.partial, 0, ctx->lay.w_partial_bytes, ctx->stream));
             CHECK(prof_begin(ctx));
-            KL(launch_transform_wide(ctx->stream, X + off * D, cnt, D, wb, &ctx->result()->status));
-            KL(launch_lse_wide(ctx->stream, cnt, D, K, wb, grid1, &ctx->result()->status));
+            KL(launch_transform_wide(ctx->stream, Xs, cnt, D, wb, &ctx->result()->status));
+            KL(launch_lse_wide(ctx->stream, cnt, D, K, wb, ctx->sms, &ctx->result()->status));
+            if (ctx->wide_refine) KL(launch_refine_wide(ctx->stream, Xs, cnt, D, K, mu, ctx->w2(), ctx->c2d(), wb));
+            else CU(cudaMemcpyAsync(wb.logz_x, wb.logz, (size_t)cnt * 8, cudaMemcpyDeviceToDevice, ctx->stream));
+            if (n_ill > 0)
+                KL(launch_lse_fp32(ctx->stream, Xs, cnt, D, n_ill, wb.mu_c, wb.w2_c, wb.c2d_c, ctx->center(), ctx->logZ2(), nullptr, wb.logz));
+            KL(launch_merge_ll_wide(ctx->stream, cnt, wb, n_ill > 0 ? ctx->logZ2() : nullptr));
             KL(launch_em_wide(ctx->stream, cnt, D, K, wb, ctx->sms, &ctx->result()->status));
             CHECK(prof_end(ctx));
             KL(launch_reduce_wide(ctx->stream, D, K, wb, ctx->sms, Nk, S1, S2));
+            if (n_ill > 0) {
+                double* Nk_c = wb.stats_c;
+                double* S1_c = Nk_c + n_ill;
+                double* S2_c = S1_c + (size_t)n_ill * D;
+                if (n_a > 0) {
+                    KL(launch_mstep_fp32(ctx->stream, Xs, cnt, D, n_a, wb.mu_c, wb.w2_c, wb.c2d_c, ctx->center(), wb.logz_x, ctx->partials(), plan_a, true));
+                    KL(launch_reduce_partials(ctx->stream, D, n_a, plan_a.splits, ctx->partials(), ctx->center(), Nk_c, S1_c, S2_c, true));
+                }
+                if (n_b > 0) {
+                    const size_t o = (size_t)n_a * D;
+                    KL(launch_mstep_fp32(ctx->stream, Xs, cnt, D, n_b, wb.mu_c + o, wb.w2_c + o, wb.c2d_c + n_a, ctx->center(), wb.logz_x, ctx->partials(), plan_b, true));
+                    KL(launch_reduce_partials(ctx->stream, D, n_b, plan_b.splits, ctx->partials(), ctx->center(), Nk_c + n_a, S1_c + o, S2_c + o, true));
+                }
+            }
         }
-        KL(launch_reduce_ll(ctx->stream, wb.llpart, grid1 < 256 ? grid1 : 256, &ctx->result()->ll[slot], true));
+        if (n_ill > 0) KL(launch_ill_scatter_wide(ctx->stream, D, K, n_ill, wb, Nk, S1, S2));
+        KL(launch_reduce_ll(ctx->stream, wb.llpart, WIDE_LL_BLOCKS, &ctx->result()->ll[slot], true));
         return GMM_OK;
     }
     if (path == GMM_PATH_TENSOR) {
@@ -533,6 +604,8 @@ int gmm_create(gmm_ctx** out, int device, void* cuda_stream) {
     if (const char* e = std::getenv("GMM_TC_COND_LIMIT")) ctx->tc_cond_limit = (float)std::atof(e);
     if (const char* e = std::getenv("GMM_TC_FILTER")) ctx->tc_force_filter = (e[0] == 't') ? 1 : (e[0] == 'p' ? 0 : -1);
     if (const char* e = std::getenv("GMM_TC_FLUSH")) ctx->tc_flush = std::atoi(e);
+    if (const char* e = std::getenv("GMM_WIDE_MIN_POINTS")) ctx->wide_min_points = std::atof(e);
+    if (const char* e = std::getenv("GMM_WIDE_REFINE")) ctx->wide_refine = std::atoi(e) != 0;
     if (const char* e = std::getenv("GMM_WIDE_PIECE")) {
         const long long v = std::atoll(e);
         if (v >= 256 && v <= WIDE_PIECE) ctx->wide_piece = v / 256 * 256;
@@ -590,6 +663,12 @@ int gmm_set_path(gmm_ctx* ctx, int path) {
 }
 
 int gmm_last_path(const gmm_ctx* ctx) { return ctx ? ctx->last_path : GMM_EINVAL; }
+
+int gmm_last_exact_count(const gmm_ctx* ctx) {
+    if (!ctx) return GMM_EINVAL;
+    if (ctx->last_path != GMM_PATH_TENSOR) return 0;
+    return wide_supports(ctx->capD, ctx->capK) ? ctx->wide_n_ill : ctx->tc_n_ill;
+}
 
 int gmm_em_step(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const float* pi, const float* mu,
                 const float* var, double* Nk, double* S1, double* S2, double* loglik) {

@@ -27,6 +27,7 @@ EXPORTS = {
     "gmm_destroy": (ctypes.c_int, [ctypes.c_void_p]),
     "gmm_set_path": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int]),
     "gmm_last_path": (ctypes.c_int, [ctypes.c_void_p]),
+    "gmm_last_exact_count": (ctypes.c_int, [ctypes.c_void_p]),
     "gmm_tensor_path_supports": (ctypes.c_int, [ctypes.c_int, ctypes.c_int]),
     "gmm_auto_path": (ctypes.c_int, [ctypes.c_int, ctypes.c_int]),
     "gmm_em_step": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_int,
@@ -192,6 +193,9 @@ class Context:
 
     def gmm_last_path(self) -> int:
         return int(lib.gmm_last_path(self._h))
+
+    def gmm_last_exact_count(self) -> int:
+        return int(lib.gmm_last_exact_count(self._h))
 
     def gmm_launch_count(self) -> int:
         return int(lib.gmm_launch_count(self._h))

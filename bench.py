@@ -156,6 +156,7 @@ def main():
 
     from paper_2606_10896_b200 import flashgmm as fg
     from paper_2606_10896_b200 import synth
+    from paper_2606_10896_b200.sharded import ShardedEM
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -187,6 +188,7 @@ def main():
     torch.cuda.synchronize()
     bytes_X = X.numel() * 4
 
+    free_before_ctx = torch.cuda.mem_get_info()[0]
     ctx = fg.Context(local)
     ctx.gmm_set_path({"auto": fg.GMM_PATH_AUTO, "fp32": fg.GMM_PATH_FP32, "tensor": fg.GMM_PATH_TENSOR}[args.path])
     pi = torch.as_tensor(pi0, device=dev)
@@ -197,19 +199,20 @@ def main():
     S2 = torch.empty((K, D), dtype=torch.float64, device=dev)
     N_global = N * world
     trace = []
+    # the sharded iteration of the package: gmm_em_step on this rank's rows, one packed all-reduce of the statistics
+    # and the log-likelihood (skipped on one GPU), replicated gmm_finalize
+    em = ShardedEM(ctx, em_step=lambda X_, p_, m_, v_: ctx.gmm_em_step(X_, p_, m_, v_, out=(Nk, S1, S2)),
+                   finalize=lambda n_, a_, b_, c_, fl_, p_, m_, v_: ctx.gmm_finalize(n_, a_, b_, c_, fl_, p_, m_, v_))
+    exact_counts = []
 
     def step():
-        _, _, _, L = ctx.gmm_em_step(X, pi, mu, var, out=(Nk, S1, S2))
-        if world > 1:
-            dist.all_reduce(Nk)
-            dist.all_reduce(S1)
-            dist.all_reduce(S2)
-        ctx.gmm_finalize(N_global, Nk, S1, S2, spec.var_floor, pi, mu, var)
-        trace.append(L)
+        trace.append(em.step(X, pi, mu, var, N_global, spec.var_floor))
+        exact_counts.append(ctx.gmm_last_exact_count())
 
     for _ in range(args.warmup):
         step()
     torch.cuda.synchronize()
+    scratch_measured = free_before_ctx - torch.cuda.mem_get_info()[0]      # everything allocated since the context was made
     if world > 1:
         dist.barrier()
     ctx.gmm_set_profiling(True)
@@ -243,35 +246,59 @@ def main():
     flops_step = 8.0 * N * K * D                      # algorithmic: two E-step and two M-step contractions
     kern_ms_step = kern_ms / args.steps
     achieved_tf = flops_step / (kern_ms_step * 1e-3) / 1e12
+    # the two secondary rates, measured now on this device (two launches of a few ms each, outside every timed region)
+    try:
+        fma_flops, ex2_rate = fg.gmm_probe_rates(local)
+    except Exception:  # noqa: BLE001
+        fma_flops, ex2_rate = 0.0, 0.0
+    wide = D > 128
     if path_used == fg.GMM_PATH_TENSOR:
         bound, peak_tf = "tensor", peaks["bf16_sustained"]
         peak_note = f"{peaks['source']} dense bf16/fp16 tensor throughput, sustained"
-        executed_factor = 24.0 / 8.0      # three fp16 products per contraction (hi*hi, hi*lo, lo*hi)
-        timed_launch = "tc_transform_kernel + em_tc_kernel per piece of 2^19 points (both inside the timed bracket)"
+        if wide:
+            executed_factor = 36.0 / 8.0  # the E-step runs in both sweeps: 3 + 3 + 3 fp16 products per pair of contractions
+            timed_launch = ("per piece of 2^17 points: wide_transform_kernel + lse_wide_kernel + em_wide_kernel, plus the FP32 "
+                            "kernels over the exactly evaluated components (all inside the timed bracket)")
+            traffic_key = "wide"
+        else:
+            executed_factor = 24.0 / 8.0      # three fp16 products per contraction (hi*hi, hi*lo, lo*hi)
+            timed_launch = "tc_transform_kernel + em_tc_kernel per piece of points (both inside the timed bracket)"
+            traffic_key = "tensor"
     else:
         bound = "alu"
-        peak_tf = 148 * 128 * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12
-        peak_note = "derived FP32 FMA peak: 148 SMs x 128 lanes x 2 flop x max SM clock"
+        if fma_flops > 0:
+            peak_tf = fma_flops / 1e12
+            peak_note = "FP32 FMA rate measured on this device by gmm_probe_rates (dependent FMA chains, full occupancy)"
+        else:
+            peak_tf = 148 * 128 * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12
+            peak_note = "derived FP32 FMA peak: 148 SMs x 128 lanes x 2 flop x max SM clock"
         executed_factor = 16.0 / 8.0
         timed_launch = "lse_kernel + M-step kernel per super-tile of 2^20 points"
-    traffic = None
+        traffic_key = "fp32_wide" if wide else "fp32"
+    # DRAM traffic of the timed kernels: bytes per point from the ncu capture summarised under profiles/ (a counter cannot
+    # be read inside an untraced run), scaled to the points of one bracketed launch
+    traffic, traffic_source = None, None
     tp = ROOT / "profiles" / "traffic.json"
     if tp.exists():
         try:
-            tj = json.loads(tp.read_text()).get("tensor" if path_used == fg.GMM_PATH_TENSOR else "fp32")
+            tj = json.loads(tp.read_text()).get(traffic_key)
             if tj:
                 traffic = tj["dram_bytes_per_point"] * N / max(1, kern_n // args.steps)
+                traffic_source = f"profiles/{tj.get('summary', 'traffic.json')}: {tj['dram_bytes_per_point']:.0f} B per point from one ncu capture, scaled by the points of a launch"
         except Exception:
             traffic = None
     roofline = {
         "bound": bound, "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved_tf / peak_tf,
-        "traffic": traffic, "peak_source": peak_note, "kernel_ms_per_step": kern_ms_step,
+        "traffic": traffic, "traffic_source": traffic_source, "peak_source": peak_note, "kernel_ms_per_step": kern_ms_step,
         "kernel_launches_per_step": kern_n / args.steps, "timed_launch": timed_launch,
         "algorithmic_flop_per_step": flops_step,
         "frac_executed": achieved_tf * executed_factor / peak_tf,
         "frac_fp32_accurate_tensor": (achieved_tf / (peak_tf / 3.0)) if bound == "tensor" else None,
         "hbm_frac": (bytes_X + 2 * K * D * 4) / (kern_ms_step * 1e-3) / 1e9 / peaks["hbm_gbs"],
-        "ex2_per_s": N * K / (kern_ms_step * 1e-3),
+        "ex2_per_s": N * K * (2 if (wide and path_used == fg.GMM_PATH_TENSOR) else 1) / (kern_ms_step * 1e-3),
+        "mufu_peak_ex2_per_s": ex2_rate or None,
+        "mufu_frac": (N * K * (2 if (wide and path_used == fg.GMM_PATH_TENSOR) else 1) / (kern_ms_step * 1e-3) / ex2_rate) if ex2_rate else None,
+        "fp32_fma_tflops_measured": (fma_flops / 1e12) if fma_flops else None,
     }
 
     # ---- optional: the top-m assignment pass over the same X, under the parameters the EM steps left ----
@@ -283,7 +310,7 @@ def main():
         ctx.gmm_assign_topm(X, pi, mu, var, m, out=(idx, resp))           # warm-up (allocates the record buffer)
         torch.cuda.synchronize()
         a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        reps = max(1, min(args.steps, 3))
+        reps = 1 if D > 128 else max(1, min(args.steps, 3))
         a0.record()
         for _ in range(reps):
             ctx.gmm_assign_topm(X, pi, mu, var, m, out=(idx, resp))
@@ -308,7 +335,7 @@ def main():
 
     # ---- optional: Fisher vectors of groups of consecutive points of the same X, under the same parameters ----
     fisher = None
-    if args.fisher_points > 0:
+    if args.fisher_points > 0 and D <= 128:          # (at D = 768, K = 4096 one vector is 25 MB: not part of this line)
         T = args.fisher_points
         n_fv = int(min(N, 2_000_000)) // T * T
         if n_fv >= T:
@@ -392,7 +419,9 @@ def main():
         line = {
             "metric": METRIC, "value": ms_step, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_step, "higher_is_better": False, "scaling": "weak", "vs_baseline": vs,
-            "dtype": "f16x2-split tensor / f32 accumulate" if path_used == fg.GMM_PATH_TENSOR else "f32",
+            "dtype": "f16" if path_used == fg.GMM_PATH_TENSOR else "f32",
+            "dtype_note": ("every operand split into two fp16 values (22 bits), three tensor-core products per contraction, fp32 "
+                           "accumulation, float64 statistics" if path_used == fg.GMM_PATH_TENSOR else "fp32 direct differences, float64 statistics"),
             "data": "synthetic",
             "config": {"workload": f"config {cfg}: N={N} per GPU, D={D}, K={K}, diagonal GMM, one EM iteration per step",
                        "path": "tensor" if path_used == fg.GMM_PATH_TENSOR else "fp32",
@@ -401,7 +430,9 @@ def main():
             "point_component_dim_per_s": N_global * K * D / (ms_step * 1e-3),
             "algorithmic_tflops": 8.0 * N_global * K * D / (ms_step * 1e-3) / 1e12,
             "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": int(launches),
-            "clocks": clocks, "scratch_bytes": int(mem_extra), "assign_topm": assign, "fisher_vectors": fisher,
+            "clocks": clocks, "scratch_bytes": int(mem_extra), "scratch_bytes_measured": int(scratch_measured),
+            "exact_components_per_step": exact_counts[-args.steps:] if exact_counts else None,
+            "assign_topm": assign, "fisher_vectors": fisher,
             "loglik_first_last": [trace[0], trace[-1]],
             "paper_context": {"A100_ms_per_iter_N1M": 3755.0 / 30, "A100_ms_per_iter_N100M": 74270.0 / 30},
         }

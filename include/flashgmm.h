@@ -263,6 +263,12 @@ int gmm_set_profiling(gmm_ctx* ctx, int on);
 int gmm_kernel_time(gmm_ctx* ctx, double* total_ms, int64_t* launches);
 int gmm_reset_counters(gmm_ctx* ctx);
 
+/* Measures, on the given device, the two rates the secondary roofs of an EM iteration are quoted against: dependent
+ * fp32 fused multiply-adds at full occupancy (in flop/s, 2 per FMA: the roof of the FP32 path) and ex2.approx.ftz.f32
+ * results per second (the special-function unit: the roof of the N K exponentials).  Two launches of a few milliseconds
+ * each on the default stream; allocates and frees 256 bytes.  Host outputs. */
+int gmm_probe_rates(int device, double* fp32_fma_flops, double* ex2_per_s);
+
 const char* gmm_strerror(int code);
 const char* gmm_last_error(const gmm_ctx* ctx);
 const char* gmm_version(void);

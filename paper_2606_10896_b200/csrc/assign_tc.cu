@@ -31,9 +31,6 @@
 
 #define TC_WAIT_LIMIT_NS 2000000000ull
 #include "tc_prims.cuh"
-#ifdef FLASHGMM_DEBUG
-#include <cstdlib>
-#endif
 
 namespace fg {
 
@@ -61,9 +58,6 @@ struct AssignParams {
     float* rec;                // [n][2][RECW] records (see assign_recw)
     int* status;
     const int* gate;           // the launch does nothing when gate[0] != 0 (too many ill-conditioned components: the FP32 kernels run instead)
-#ifdef FLASHGMM_DEBUG
-    int dbg;                   // what-if timing only (results are wrong): 1 no selection, 2 no softmax arithmetic, 4 no MMAs, 8 no B loads
-#endif
 };
 
 constexpr int assign_recw(int LIST) { return (2 + 2 * LIST + 3) & ~3; }      // words per record: m, s, LIST values, LIST indices
@@ -138,9 +132,6 @@ assign_tc_kernel(const AssignParams p, const __grid_constant__ CUtensorMap tm_yh
                         fence_before();
                         bar_arrive(BAR(AB_LEMPTY + grp));
                     }
-#ifdef FLASHGMM_DEBUG
-                    if (p.dbg & 2) continue;
-#endif
                     const int col0 = c * AT_COMPS + sub * 32;
                     const float4* tc4 = reinterpret_cast<const float4*>(p.tkck + col0);
                     float l[32];
@@ -164,9 +155,6 @@ assign_tc_kernel(const AssignParams p, const __grid_constant__ CUtensorMap tm_yh
                     }
                     s_run += acc0 + acc1;
                     // the LIST largest: most blocks hold nothing that beats any lane's current LIST-th value
-#ifdef FLASHGMM_DEBUG
-                    if (p.dbg & 1) continue;
-#endif
                     if (__any_sync(0xffffffffu, bmax > tv[LIST - 1])) {
 #pragma unroll
                         for (int j = 0; j < 32; ++j) {
@@ -235,16 +223,9 @@ assign_tc_kernel(const AssignParams p, const __grid_constant__ CUtensorMap tm_yh
                     if (use > 0 && !wait0(BAR(AB_BEMPTY + st), (uint32_t)((use - 1) & 1))) { ok = false; break; }
                     if (elect_one()) {
                         const uint32_t dst = smem_u32(smem + ASM_B + st * 2 * AT_ATOM);
-#ifdef FLASHGMM_DEBUG
-                        if (p.dbg & 8) bar_arrive(BAR(AB_BFULL + st));
-                        else {
-#endif
                         bar_expect_tx(BAR(AB_BFULL + st), 2 * AT_ATOM);
                         tma_load_3d(dst, &tm_phi, 0, c * AT_COMPS, a, BAR(AB_BFULL + st));
                         tma_load_3d(dst + AT_ATOM, &tm_plo, 0, c * AT_COMPS, a, BAR(AB_BFULL + st));
-#ifdef FLASHGMM_DEBUG
-                        }
-#endif
                     }
                     __syncwarp();
                     ++g;
@@ -294,9 +275,6 @@ assign_tc_kernel(const AssignParams p, const __grid_constant__ CUtensorMap tm_yh
                         const uint64_t ah = d_ahi + ((a * AT_ATOM) >> 4), al = d_alo + ((a * AT_ATOM) >> 4);
                         const uint64_t bh = d_b + ((st * 2 * AT_ATOM) >> 4), bl = bh + (AT_ATOM >> 4);
                         // the two small cross products first, then the leading one (as in the E-step of the tile kernel)
-#ifdef FLASHGMM_DEBUG
-                        if (!(p.dbg & 4)) {
-#endif
 #pragma unroll
                         for (int j = 0; j < 4; ++j)
                             if (j < kk) mma_ss(d, ah + ((j * 32) >> 4), bl + ((j * 32) >> 4), idesc, (a > 0 || j > 0) ? 1u : 0u);
@@ -306,9 +284,6 @@ assign_tc_kernel(const AssignParams p, const __grid_constant__ CUtensorMap tm_yh
 #pragma unroll
                         for (int j = 0; j < 4; ++j)
                             if (j < kk) mma_ss(d, ah + ((j * 32) >> 4), bh + ((j * 32) >> 4), idesc, 1u);
-#ifdef FLASHGMM_DEBUG
-                        }
-#endif
                         mma_commit(BAR(AB_BEMPTY + st));
                         if (c == NC - 1) mma_commit(BAR(AB_AEMPTY + a));
                         if (a == n_atoms - 1) mma_commit(BAR(AB_LFULL + b));
@@ -398,12 +373,6 @@ struct PointRow {
     }
 };
 
-#ifdef FLASHGMM_DEBUG
-__device__ unsigned long long g_refine_counts[4];     // points answered by one thread, exact candidate evaluations, exact ill evaluations, rows left uncertain
-#define RCOUNT(i, v) do { if (lane == 0) atomicAdd(&g_refine_counts[i], (unsigned long long)(v)); } while (0)
-#else
-#define RCOUNT(i, v)
-#endif
 
 // Warp-uniform list (every lane holds the same copy) of the MAXM largest exact values seen so far: descending, equal
 // values in ascending component order, whatever the order of insertion.
@@ -520,7 +489,6 @@ __device__ __forceinline__ void refine_point(const RefineArgs& g, const TcIllCac
                 alive_set &= alive_set - 1;
                 float mag;
                 const float e = __ldg(g.c2 + k) - pr.quad<false>(g.mu + (size_t)k * D, g.w2 + (size_t)k * D, D, lane, mag);
-                RCOUNT(2, 1);
                 if (e > NEG) {
                     top.insert(e, k);
                     ++n_exact;
@@ -564,7 +532,6 @@ __device__ __forceinline__ void refine_point(const RefineArgs& g, const TcIllCac
         for (int r = 0; r < C; ++r) {
             if (r < p) {
                 const float e = __ldg(g.c2 + kv[r]) - qv[r];
-                RCOUNT(1, 1);
                 if (lane == r) { ev = e; ea = sv; }
                 if (e > NEG) { top.insert(e, kv[r]); ++n_exact; }
             }
@@ -612,7 +579,6 @@ __device__ __forceinline__ void refine_point(const RefineArgs& g, const TcIllCac
         }
         return;
     }
-    RCOUNT(3, 1);
     // Not certain (near ties, exact ties, too few finite candidates, broad posteriors): the point joins the list of rows
     // that the FP32 tile kernel evaluates against all K components afterwards.  (The order of the list varies from run to
     // run; the result of a row does not depend on it.)
@@ -709,9 +675,6 @@ assign_refine_kernel(const float* __restrict__ rec, const float* __restrict__ X,
                     if (resp_out) resp_out[row * m + j] = __fdividef(fast_ex2(al.a[j] - M), S);
                 }
             }
-#ifdef FLASHGMM_DEBUG
-            atomicAdd(&g_refine_counts[0], 1ull);
-#endif
         }
         unsigned todo = __ballot_sync(0xffffffffu, valid && !sharp);
         while (todo) {
@@ -741,9 +704,6 @@ cudaError_t launch_assign_t(cudaStream_t s, const float* X, int64_t n, int D, in
     p.n = n; p.n_chunks = pl.CL; p.n_ks = pl.n_ks;
     p.tkck = reinterpret_cast<const float2*>(tb.tkck);
     p.rec = rec; p.status = status; p.gate = tb.flags + 3;
-#ifdef FLASHGMM_DEBUG
-    p.dbg = std::getenv("GMM_AT_DBG") ? std::atoi(std::getenv("GMM_AT_DBG")) : 0;
-#endif
     const int64_t rows_padded = (n + TC_BN - 1) / TC_BN * TC_BN;       // what launch_transform_tc wrote
     CUtensorMap tm_yhi, tm_ylo, tm_phi, tm_plo;
     cudaError_t e = tc_make_plane_map(&tm_yhi, tb.y_hi, rows_padded, AT_POINTS, 1);
@@ -776,13 +736,6 @@ cudaError_t launch_assign_t(cudaStream_t s, const float* X, int64_t n, int D, in
 
 }  // namespace
 
-#ifdef FLASHGMM_DEBUG
-extern "C" void gmm_debug_refine_counts(unsigned long long* out) {
-    cudaMemcpyFromSymbol(out, g_refine_counts, sizeof(g_refine_counts));
-    unsigned long long z[4] = {0, 0, 0, 0};
-    cudaMemcpyToSymbol(g_refine_counts, z, sizeof(z));
-}
-#endif
 
 // LIST = 6 (m <= 4) or 10: the m wanted, at least one spare candidate, and the best value left outside (for the certainty
 // test).  Small m keeps 5 candidates too: the responsibilities are only as accurate as the share of the log-sum-exp that

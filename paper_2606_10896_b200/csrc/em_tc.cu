@@ -31,9 +31,6 @@
 
 #include <cuda.h>
 #include <cuda_fp16.h>
-#ifdef FLASHGMM_DEBUG
-#include <cstdio>
-#endif
 #include <math_constants.h>
 
 namespace fg {
@@ -74,15 +71,6 @@ constexpr int SMEM_BYTES = SM_END + 1024;       // + alignment slack
 enum { B_YFULL0 = 0, B_YFULL1, B_YEMPTY0, B_YEMPTY1, B_LFULL0, B_LFULL1, B_RREADY0, B_RREADY1, B_ACCFULL,
        B_ACCFREE, B_FINAL, B_COUNT };
 
-#ifdef FLASHGMM_DEBUG
-#define TIC(var) long long var = clock64()
-#define TOC(var, slot) do { if (p.dbg_clk && blockIdx.x == 0) { long long now_ = clock64(); if ((threadIdx.x & 31) == 0) atomicAdd((unsigned long long*)&p.dbg_clk[slot], (unsigned long long)(now_ - var)); var = now_; } } while (0)
-#define TRACE(ev, tile) do { if (p.dbg_trace && blockIdx.x == 0 && (tile) < 64) p.dbg_trace[(tile) * 16 + (ev)] = clock64(); } while (0)
-#else
-#define TIC(var)
-#define TOC(var, slot)
-#define TRACE(ev, tile)
-#endif
 
 // ---- exchange between the CTAs of a group through global memory (L2).  A slot is two 64-bit words {value, tag}: each
 //      word is written and read as one unit, so a reader that sees the expected tag in both words has both values.
@@ -244,13 +232,6 @@ struct TcKernelParams {
     // points (0 .. BN; the rest of its rows are zeros) taken from rows tile_src[t] .. of X.  Both NULL otherwise.
     const int* tile_valid;
     const int64_t* tile_src;
-#ifdef FLASHGMM_DEBUG
-    float* dbg;      // [Kpad][64] log2 z of the first tile
-    int dbg_cluster, dbg_i; // which (group, local tile) the logit dump records
-    uint4* dbg_y;           // [4096] copy of the Y stage as the issuer finds it after its wait (CTA rank 0 of the group)
-    long long* dbg_clk;   // per-phase cycle counters of CTA 0
-    long long* dbg_trace; // [64 tiles][16 events] clock64 stamps of CTA 0
-#endif
 };
 
 // BIG: groups of more than 8 CTAs (1024 < K <= 4096).  TIGHT: the filter for launches in which many components are
@@ -375,27 +356,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
             const int nvalid = tile_points - p0;                                      // valid points of this group's half
             const int64_t xrow0 = p.tile_src ? __ldg(p.tile_src + tile) : row0;       // where the tile's points sit in X
 
-            TIC(tk_);
             if (!bar_wait(BAR(B_LFULL0 + s), ph, abort_flag, p.status, false)) alive = false;
-            TOC(tk_, 0);
-            if (gtid == 0) TRACE(grp ? 14 : 0, i);
             fence_after();
-#ifdef FLASHGMM_DEBUG
-            if (p.order & 4) {                // what-if timing only: no softmax work at all
-                fence_before();
-                bar_arrive(BAR(B_RREADY0 + s));
-                const bool pe = (i & 1) || (i + 1 == ntl);
-                const int64_t pn = (i | 1) + 1;
-                if (grp == 1 && pe && ((pn % p.flush) == 0 || pn >= ntl)) {
-                    const uint32_t fpar = (uint32_t)(((pn - 1) / p.flush) & 1);
-                    bar_wait(BAR(B_ACCFULL), fpar, abort_flag, p.status, false);
-                    fence_after();
-                    fence_before();
-                    bar_arrive(BAR(B_ACCFREE));
-                }
-                continue;
-            }
-#endif
             float l[32];
             {
                 uint32_t v0[32];
@@ -404,11 +366,6 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
 #pragma unroll
                 for (int j = 0; j < 32; ++j) l[j] = fmaf(__uint_as_float(v0[j]), tk, ck);
             }
-#ifdef FLASHGMM_DEBUG
-            if (p.dbg && cluster_id == p.dbg_cluster && i == p.dbg_i)
-                for (int j = 0; j < 32; ++j) p.dbg[(size_t)(rank * 128 + kloc) * 64 + p0 + j] = l[j];
-#endif
-            TOC(tk_, 16);
             float red;
             // Ill-conditioned components (sum_d mu^2 / var too large for the 22-bit expanded form, e.g. a component
             // collapsed onto one point at the variance floor): their approximate logits carry an error of up to E_k.
@@ -441,10 +398,6 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                 const float lb_own = tight ? red : red - emax_w;
                 uint32_t mlo = 0;
                 if (emax_w > 0.f) {
-#ifdef FLASHGMM_DEBUG
-                    if (p.dbg_clk && blockIdx.x == 0 && lane == 0) atomicAdd((unsigned long long*)&p.dbg_clk[26], 1ull);
-                    if (p.dbg_clk && blockIdx.x == 0 && i == 0 && illb > 0.f) atomicAdd((unsigned long long*)&p.dbg_clk[27], 1ull);
-#endif
                     // Local filter, by shuffles (no shared memory, no warp barrier: a barrier here would also wait for
                     // global stores in flight): bit j of mlo = point j of this lane's component may matter.
                     // (only flagged lanes: in the tight mode a warp without a well-conditioned component has the bound -inf,
@@ -504,12 +457,10 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                 // publish AFTER the filter: peers read these slots only for the rare pairs that survive their own filter,
                 // and a global store in flight makes the next warp-level barrier wait for it
                 xslot_write(ring + (rank * 4 + wq) * 64 + lane, lb_own, 0.f, tag);
-                TOC(tk_, 28);
                 if (emax_w > 0.f) {
                     const int kglob = (int)rank * 128 + kloc;
                     bool fixed_any = false;
                     uint32_t exact_mask = 0;                                 // points of this lane's component recomputed exactly
-                    TOC(tk_, 29);
                     // Second filter, against the GROUP-wide lower bound of each point (the maximum of the bounds that all
                     // 4 CL warps of the group published).  That bound depends on the point only, so it is fetched once per
                     // point that has candidates - four points per L2 round trip, lane c reading the slot of
@@ -520,10 +471,6 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                     uint32_t pm = have_cand ? __reduce_or_sync(0xffffffffu, mlo) : 0u;       // points with at least one candidate
                     float lb_keep = CUDART_INF_F;                            // lane j keeps the group bound of point j
                     while (pm != 0u && alive) {
-#ifdef FLASHGMM_DEBUG
-                        if (p.dbg_clk && blockIdx.x == 0 && lane == 0) atomicAdd((unsigned long long*)&p.dbg_clk[24], 1ull);
-                        if (p.dbg_clk && blockIdx.x == 0 && lane == 0) atomicAdd((unsigned long long*)&p.dbg_clk[23], (unsigned long long)__popc(pm));
-#endif
                         int jb[4];
                         uint32_t rest = pm;
 #pragma unroll
@@ -587,9 +534,6 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                         int j = __ffs(mlo) - 1;
                         j = __shfl_sync(0xffffffffu, j, src);
                         const int kk = __shfl_sync(0xffffffffu, kglob, src);
-#ifdef FLASHGMM_DEBUG
-                        if (p.dbg_clk && blockIdx.x == 0 && lane == 0) atomicAdd((unsigned long long*)&p.dbg_clk[25], 1ull);
-#endif
                         const float* xr = p.X + (xrow0 + p0 + j) * p.D;
                         const float* mr = p.mu + (size_t)kk * p.D;
                         const float* wr = p.w2 + (size_t)kk * p.D;
@@ -619,14 +563,12 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                             if (!((exact_mask >> jj) & 1u)) l[jj] = -CUDART_INF_F;
                     }
                     __syncwarp();
-                    TOC(tk_, 30);
                     if (fixed_any) warp_reduce_scatter32<true>(l, red, lane);      // maxima with the corrected logits
                 }
             }
             // all-gather the warp maxima through shared memory
             gather[lane] = red;
             __syncwarp();
-            TOC(tk_, 17);
 #pragma unroll
             for (int j = 0; j < 32; j += 4) {
                 const float4 m4 = *reinterpret_cast<const float4*>(gather + j);
@@ -640,14 +582,10 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                 l[j + 3] = fast_ex2(l[j + 3] - m3);
             }
             __syncwarp();
-            TOC(tk_, 18);
             float sred;
             warp_reduce_scatter32<false>(l, sred, lane);
             ws[wq * 32 + lane] = make_float2(red, sred);
-            TOC(tk_, 1);
             named_bar_sync(1 + 2 * grp, 128);
-            TOC(tk_, 2);
-            if (gtid == 0) TRACE(1, i);
             if (gtid < 32) {
                 const int pt = gtid;
                 float2 w4[4];
@@ -664,46 +602,30 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                 XSlot* ring = xg + (size_t)(i & 3) * p.CL * 64 + p0 + pt;
                 // (test hook: one CTA stays silent for the first tile, so that its peers' bounded waits run out)
                 if (!(p.test_silent_rank == (int)rank && cluster_id == 0 && i == 0)) xslot_write(ring + rank * 64, mc, sc, tag);
-                TOC(tk_, 3);
                 float mi = -CUDART_INF_F, mi_safe = 0.f, Z = 0.f;
                 if (!BIG) {
                     float2 e[8];
-#ifdef FLASHGMM_DEBUG
-                    if (p.order & 64) {           // what-if timing only (results are wrong): do not wait for the peers
-#pragma unroll
-                        for (int c = 0; c < 8; ++c) e[c] = make_float2(mc, sc);
-                    } else
-#endif
                     if (!xslot_wait_all(ring, p.CL, tag, e, abort_flag, p.status)) alive = false;
 #pragma unroll
                     for (int c = 0; c < 8; ++c) mi = fmaxf(mi, e[c].x);
-                    TOC(tk_, 4);
-                    if (gtid == 0) TRACE(2, i);
                     mi_safe = (mi == -CUDART_INF_F) ? 0.f : mi;
 #pragma unroll
                     for (int c = 0; c < 8; ++c)
                         Z += (e[c].x == -CUDART_INF_F) ? 0.f : e[c].y * fast_ex2(e[c].x - mi_safe);
                 } else {
                     if (!xslot_collect_many(ring, p.CL, tag, mi, Z, abort_flag, p.status)) alive = false;
-                    TOC(tk_, 4);
-                    if (gtid == 0) TRACE(2, i);
                     mi_safe = (mi == -CUDART_INF_F) ? 0.f : mi;
                 }
-                TOC(tk_, 19);
                 const bool valid = pt < nvalid;
                 const float inv = (valid && Z > 0.f) ? __fdividef(RSCALE, Z) : 0.f;
 #pragma unroll
                 for (int w = 0; w < 4; ++w)
                     fac[w * 32 + pt] = (w4[w].x == -CUDART_INF_F) ? 0.f : fast_ex2(w4[w].x - mi_safe) * inv;
-                TOC(tk_, 20);
                 ll_have = rank == 0 && valid;
                 ll_m = mi; ll_z = Z;
             }
             if (gtid == 0) decision_s[grp] = *abort_flag;
-            TOC(tk_, 5);
             named_bar_sync(2 + 2 * grp, 128);
-            TOC(tk_, 6);
-            if (gtid == 0) TRACE(3, i);
             if (decision_s[grp]) break;
             // responsibilities: r = p * fac, split into fp16 hi + lo, written over the logits as the M-step A operand
             {
@@ -735,8 +657,6 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
             }
             fence_before();
             bar_arrive(BAR(B_RREADY0 + s));
-            TOC(tk_, 7);
-            if (gtid == 0) TRACE(grp ? 15 : 4, i);
             if (gtid < 32 && ll_have) {              // two-sum: (ll_s, ll_c) += log2 Z_i exactly to fp32 pair precision
                 const float v = ll_m + log2f(ll_z);
                 const float t = ll_s + v;
@@ -763,7 +683,6 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                 }
                 fence_before();
                 bar_arrive(BAR(B_ACCFREE));
-                TOC(tk_, 8);
             }
             // N_k of this group's points has its own column
             if (((i + 1) % 64) == 0 || i + 1 >= ntl) {
@@ -794,28 +713,18 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
             const int s = (int)(i & 1);
             const uint32_t ph = (uint32_t)((i >> 1) & 1);
             const int32_t row0 = (int32_t)((cluster_id + i * p.Q) * BN);
-            TIC(tt_);
             if (i >= 2) {
                 uint32_t w = 1;
                 if (lane == 0) w = bar_wait(BAR(B_YEMPTY0 + s), ph ^ 1, abort_flag, p.status, false) ? 1u : 0u;
                 w = __shfl_sync(0xffffffffu, w, 0);
                 if (!w) { ok = false; break; }
             }
-            TOC(tt_, 10);
-            if (tid == PRODUCER_WARP * 32) TRACE(5, i);
             if (elect_one()) {
                 const uint32_t bar = BAR(B_YFULL0 + s);
                 const uint32_t dst = smem_u32(smem + SM_Y + s * SM_YSTAGE);
-#ifdef FLASHGMM_DEBUG
-                if (p.order & 8) bar_arrive(bar);          // what-if timing only: no loads, the stage keeps what it holds
-                else {
-#endif
                 bar_expect_tx(bar, stage_bytes);
                 tma_load_3d(dst, &tm_hi, 0, row0, 0, bar);                 // box = (128 bytes, 64 points, n_atoms atoms)
                 tma_load_3d(dst + SM_YLO, &tm_lo, 0, row0, 0, bar);
-#ifdef FLASHGMM_DEBUG
-                }
-#endif
                 // The planes were written by another kernel and are larger than L2: ask for the tile this CTA will load
                 // two steps from now (the next one is already in flight for the other stage); one CTA of the group asks
                 // for all, in turn.
@@ -827,8 +736,6 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
             }
             __syncwarp();
             issued = i + 1;
-            TOC(tt_, 11);
-            if (tid == PRODUCER_WARP * 32) TRACE(6, i);
         }
         // On an abort the consumer may never wait for the last loads: they must have landed before the CTA may exit.
         if (!ok || *abort_flag) {
@@ -861,21 +768,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
         auto issue_E = [&](int64_t i, bool seen = false) -> bool {
             const int s = (int)(i & 1);
             const uint32_t ph = (uint32_t)((i >> 1) & 1);
-            TIC(tm_);
             if (!seen && !wait_all(BAR(B_YFULL0 + s), ph)) return false;
-            TOC(tm_, 12);
-            TRACE(7, i);
             if (elect_one()) {
-#ifdef FLASHGMM_DEBUG
-                if (p.dbg_y && rank == 0 && cluster_id == p.dbg_cluster && i == p.dbg_i) {
-                    const uint4* ys = reinterpret_cast<const uint4*>(smem + SM_Y + s * SM_YSTAGE);
-                    for (int q = 0; q < 4096; ++q) p.dbg_y[q] = ys[q];
-                }
-#endif
                 const uint32_t d = T_LOG + s * 64;
-#ifdef FLASHGMM_DEBUG
-                if (!(p.order & 16)) {        // what-if timing only: no E-step MMAs
-#endif
                 const uint64_t dyh = make_desc(y0 + s * SM_YSTAGE, 16, 1024);            // K-major views of the stage
                 const uint64_t dyl = make_desc(y0 + s * SM_YSTAGE + SM_YLO, 16, 1024);
                 // The two small cross products go first: the accumulator truncates (toward zero) at every add, by up to
@@ -884,38 +779,24 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
                 for (int ks = 0; ks < 16; ++ks)
                     if (ks < n_ks) mma_ss(d, d_plo + (((ks >> 2) * 16384 + (ks & 3) * 32) >> 4),
                                           dyh + (((ks >> 2) * 8192 + (ks & 3) * 32) >> 4), id_e, ks > 0);
-                TRACE(11, i);
 #pragma unroll
                 for (int ks = 0; ks < 16; ++ks)
                     if (ks < n_ks) mma_ts(d, T_PHI + ks * 8, dyl + (((ks >> 2) * 8192 + (ks & 3) * 32) >> 4), id_e, 1);
-                TRACE(12, i);
 #pragma unroll
                 for (int ks = 0; ks < 16; ++ks)
                     if (ks < n_ks) mma_ts(d, T_PHI + ks * 8, dyh + (((ks >> 2) * 8192 + (ks & 3) * 32) >> 4), id_e, 1);
-                TRACE(13, i);
-#ifdef FLASHGMM_DEBUG
-                }
-#endif
                 mma_commit(BAR(B_LFULL0 + s));
             }
             __syncwarp();
-            TOC(tm_, 13);
-            TRACE(8, i);
             return true;
         };
         auto issue_M = [&](int64_t i, bool seen = false) -> bool {
             const int s = (int)(i & 1);
             const uint32_t ph = (uint32_t)((i >> 1) & 1);
-            TIC(tm_);
             if (!seen && !wait_all(BAR(B_RREADY0 + s), ph)) return false;
-            TOC(tm_, 14);
-            TRACE(9, i);
             if (elect_one()) {
                 // A operand layout in the logits buffer: points 0-31 -> columns [0,16) r_hi, [16,32) r_lo; points 32-63 -> +32
                 const uint32_t rbase = T_LOG + s * 64;
-#ifdef FLASHGMM_DEBUG
-                if (!(p.order & 32)) {        // what-if timing only: no M-step MMAs
-#endif
                 const uint64_t dyh = make_desc(y0 + s * SM_YSTAGE, 8192, 1024);          // MN-major views of the stage
                 const uint64_t dyl = make_desc(y0 + s * SM_YSTAGE + SM_YLO, 8192, 1024);
 #pragma unroll
@@ -927,15 +808,10 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
 #pragma unroll
                 for (int ks = 0; ks < BN / 16; ++ks)
                     mma_ts(T_ACC, rbase + (ks >> 1) * 32 + (ks & 1) * 8 + 16, dyh + ((ks * 2048) >> 4), id_m, 1);
-#ifdef FLASHGMM_DEBUG
-                }
-#endif
                 mma_commit(BAR(B_YEMPTY0 + s));
             }
             __syncwarp();
             acc_valid = true;
-            TOC(tm_, 15);
-            TRACE(10, i);
             return true;
         };
         // Hands the TMEM accumulators to the flushing softmax group and waits until they are free again.
@@ -1028,19 +904,6 @@ __global__ void __launch_bounds__(NTHREADS, 1) em_tc_kernel(const TcKernelParams
     // teardown: everybody meets, peers are done with this CTA's shared memory, TMEM is released
     fence_before();
     __syncthreads();
-#ifdef FLASHGMM_DEBUG
-    if (p.dbg) {       // is the P_lo image in shared memory still what the prologue copied?
-        const uint4* src = reinterpret_cast<const uint4*>(p.plo_img + (size_t)rank * 65536);
-        const uint4* dst = reinterpret_cast<const uint4*>(smem + SM_PLO);
-        int bad = 0, first = -1;
-        for (int i = tid; i < 65536 / 16; i += NTHREADS) {
-            const uint4 a = __ldg(src + i), b = dst[i];
-            if (a.x != b.x || a.y != b.y || a.z != b.z || a.w != b.w) { ++bad; if (first < 0) first = i; }
-        }
-        if (bad && blockIdx.x < 8) printf("CTA %d thread %d: %d P_lo chunks differ, first chunk %d\n", (int)blockIdx.x, tid, bad, first);
-    }
-    __syncthreads();
-#endif
     if (warp == MMA_WARP) {
         fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512) : "memory");
@@ -1549,18 +1412,6 @@ cudaError_t launch_transform_grouped_tc(cudaStream_t s, const float* X, int64_t 
     return cudaGetLastError();
 }
 
-#ifdef FLASHGMM_DEBUG
-float* g_tc_debug = nullptr;
-long long* g_tc_clk = nullptr;
-long long* g_tc_trace = nullptr;
-extern "C" void gmm_debug_set_trace(long long* p) { g_tc_trace = p; }
-extern "C" void gmm_debug_set_buffer(float* p) { g_tc_debug = p; }
-int g_tc_dbg_cluster = 0, g_tc_dbg_i = 0;
-uint4* g_tc_dbg_y = nullptr;
-extern "C" void gmm_debug_set_ybuf(void* p) { g_tc_dbg_y = static_cast<uint4*>(p); }
-extern "C" void gmm_debug_set_select(int cluster, int i) { g_tc_dbg_cluster = cluster; g_tc_dbg_i = i; }
-extern "C" void gmm_debug_set_clk(long long* p) { g_tc_clk = p; }
-#endif
 
 int g_tc_order = 2;
 // test hooks of the time-out path (see tc_set_test_hooks)
@@ -1680,12 +1531,6 @@ cudaError_t launch_em_tc(cudaStream_t s, const float* X, int64_t n, int D, int K
     p.dec_dim = tb.dec_dim; p.dec_w = tb.dec_w; p.dec_mu = tb.dec_mu;
     p.partial = tb.partial; p.llpart = tb.llpart; p.status = status;
     p.xg = static_cast<XSlot*>(tb.xg); p.xl = static_cast<XSlot*>(tb.xl);
-#ifdef FLASHGMM_DEBUG
-    p.dbg = g_tc_debug;
-    p.dbg_cluster = g_tc_dbg_cluster; p.dbg_i = g_tc_dbg_i; p.dbg_y = g_tc_dbg_y;
-    p.dbg_clk = g_tc_clk;
-    p.dbg_trace = g_tc_trace;
-#endif
     cudaError_t e = set_smem_attr(big, tight);
     if (e != cudaSuccess) return e;
     // exchange slots carry the tile number as their tag: clear what the previous launch left behind

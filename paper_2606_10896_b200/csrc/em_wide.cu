@@ -687,61 +687,83 @@ __global__ void __launch_bounds__(256) wide_transform_kernel(const float* __rest
 // ------------------------------------------------------------------------------------------------------------------
 // Parameter preparation (float64 arithmetic on K * D elements).
 // One block per dimension: centre g_d = sum_k pi_k mu_kd / sum_k pi_k, scale s_d = 2^-round(log2 rms_d) with
-// rms_d^2 = sum_k pi_k ((mu_kd - g_d)^2 + var_kd), and kap_d = s_d^2 sum_k pi_k ((mu_kd - g_d)^2 - var_kd): with that
-// constant a component's own points (x = mu + sigma z) give the term a u + b (u^2 + kap) of dimension d the expectation
-// w (mu'^2 - var) / 2 - w kap / (2 s^2), which vanishes on average over the mixture, so the contraction's partial sums are a
-// zero-mean walk over the dimensions instead of growing like D / 2.
+// rms_d^2 = sum_k pi_k ((mu_kd - g_d)^2 + var_kd), and the constant kap_d added to the squares.
+// kap_d: a point of component k (x = mu + sigma z) adds a u + b (u^2 + kap) = w2 ((mu'^2 - kap') - (x' - mu')^2) to the
+// accumulator in dimension d (w2 = log2 e / (2 var), primes: centred, unscaled), on average w2 (mu'^2 - var - kap').
+// kap'_d is chosen so that this average vanishes over the mixture, each component weighted by pi_k w2_kd:
+//     kap'_d = sum_k pi_k w2_kd (mu'_kd^2 - var_kd) / sum_k pi_k w2_kd
+// (the weight w2 matters: with variances that differ between components, E[var] E[1 / var] > 1, and the plain average
+// leaves every component a drift of hundreds of log2 units at D = 768).  The contraction's partial sums are then a
+// zero-mean walk over the dimensions, tens in size instead of D / 2, and the truncation error of the tensor core's fp32
+// accumulation shrinks with them.  A component much narrower than the rest (one collapsed onto a point, say) has its
+// weight capped at 16 times that of the average variance, so that it cannot pull kap_d toward itself.
 __global__ void __launch_bounds__(128) wide_scale_kernel(int D, int K, const float* __restrict__ pi, const float* __restrict__ mu,
                                                          const float* __restrict__ var, float* __restrict__ sd,
                                                          float* __restrict__ kap, float* __restrict__ gd) {
     const int d = blockIdx.x, t = threadIdx.x;
     __shared__ double r_a[128], r_b[128], r_w[128];
-    __shared__ double g_s;
-    double a = 0.0, w = 0.0;
+    __shared__ double g_s, v_s;
+    double a = 0.0, w = 0.0, v0 = 0.0;
     if (d < D)
         for (int k = t; k < K; k += 128) {
             const double pk = (double)pi[k];
             a += pk * (double)mu[(size_t)k * D + d];
+            v0 += pk * (double)var[(size_t)k * D + d];
             w += pk;
         }
-    r_a[t] = a; r_w[t] = w;
-    __syncthreads();
-    for (int o = 64; o > 0; o >>= 1) {
-        if (t < o) { r_a[t] += r_a[t + o]; r_w[t] += r_w[t + o]; }
-        __syncthreads();
-    }
-    if (t == 0) {
-        const float gf = (r_w[0] > 0.0) ? (float)(r_a[0] / r_w[0]) : 0.f;
-        g_s = (d < D && isfinite(gf)) ? (double)gf : 0.0;
-    }
-    __syncthreads();
-    const double g = g_s;
-    double m2 = 0.0, v = 0.0;
-    w = 0.0;
-    if (d < D)
-        for (int k = t; k < K; k += 128) {
-            const double pk = (double)pi[k];
-            const double m = (double)mu[(size_t)k * D + d] - g;
-            m2 += pk * m * m;
-            v += pk * (double)var[(size_t)k * D + d];
-            w += pk;
-        }
-    __syncthreads();
-    r_a[t] = m2; r_b[t] = v; r_w[t] = w;
+    r_a[t] = a; r_b[t] = v0; r_w[t] = w;
     __syncthreads();
     for (int o = 64; o > 0; o >>= 1) {
         if (t < o) { r_a[t] += r_a[t + o]; r_b[t] += r_b[t + o]; r_w[t] += r_w[t + o]; }
         __syncthreads();
     }
     if (t == 0) {
+        const float gf = (r_w[0] > 0.0) ? (float)(r_a[0] / r_w[0]) : 0.f;
+        g_s = (d < D && isfinite(gf)) ? (double)gf : 0.0;
+        v_s = (r_w[0] > 0.0) ? r_b[0] / r_w[0] : 0.0;          // the mixture's average variance in this dimension
+    }
+    __syncthreads();
+    const double g = g_s, vbar = v_s;
+    const double wcap = (vbar > 0.0 && isfinite(vbar)) ? 16.0 / vbar : 0.0;
+    double m2 = 0.0, num = 0.0, den = 0.0;
+    w = 0.0;
+    if (d < D)
+        for (int k = t; k < K; k += 128) {
+            const double pk = (double)pi[k];
+            const double m = (double)mu[(size_t)k * D + d] - g;
+            const double v = (double)var[(size_t)k * D + d];
+            m2 += pk * m * m;
+            w += pk;
+            if (v > 0.0) {
+                const double wk = pk * fmin(1.0 / v, wcap);
+                num += wk * (m * m - v);
+                den += wk;
+            }
+        }
+    __syncthreads();
+    r_a[t] = m2; r_w[t] = w;
+    __syncthreads();
+    for (int o = 64; o > 0; o >>= 1) {
+        if (t < o) { r_a[t] += r_a[t + o]; r_w[t] += r_w[t + o]; }
+        __syncthreads();
+    }
+    const double mm_tot = r_a[0], w_tot = r_w[0];
+    __syncthreads();
+    r_a[t] = num; r_b[t] = den;
+    __syncthreads();
+    for (int o = 64; o > 0; o >>= 1) {
+        if (t < o) { r_a[t] += r_a[t + o]; r_b[t] += r_b[t + o]; }
+        __syncthreads();
+    }
+    if (t == 0) {
         float s = 1.f, kp = 0.f;
-        double mm = r_a[0], vv = r_b[0];
-        if (r_w[0] > 0.0) { mm /= r_w[0]; vv /= r_w[0]; }
-        const double ms = mm + vv;
+        const double mm = w_tot > 0.0 ? mm_tot / w_tot : 0.0;
+        const double ms = mm + vbar;
         if (d < D && ms > 0.0 && isfinite(ms)) {
             const double e = rint(0.5 * log2(ms));
             s = (float)exp2(-fmin(fmax(e, -60.0), 60.0));
-            kp = (float)((mm - vv) * (double)s * (double)s);
+            const double kq = (r_b[0] > 0.0) ? r_a[0] / r_b[0] : (mm - vbar);
+            kp = isfinite(kq) ? (float)(kq * (double)s * (double)s) : 0.f;
         }
         sd[d] = s;
         kap[d] = kp;
@@ -758,9 +780,9 @@ __global__ void __launch_bounds__(256) wide_prepare_kernel(int D, int Dpad, int 
                                                            double* __restrict__ ckd, float* __restrict__ illb,
                                                            float cond_limit, float min_weight, int* __restrict__ flags) {
     extern __shared__ double ab_s[];                     // [2][Dpad]: a, b of this component
-    __shared__ double red[4][256];
+    __shared__ double red[5][256];
     const int k = blockIdx.x, t = threadIdx.x;
-    double mx = 0.0, csum = 0.0, cond2 = 0.0;
+    double mx = 0.0, csum = 0.0, cond2 = 0.0, ramp = 0.0;
     for (int d = t; d < Dpad; d += 256) {
         double a = 0.0, b = 0.0;
         if (k < K && d < D) {
@@ -771,18 +793,21 @@ __global__ void __launch_bounds__(256) wide_prepare_kernel(int D, int Dpad, int 
             csum += m * m / v + log(6.283185307179586476925286766559 * v);
             const double tau = 0.5 * w * 3.0 * (m * m + 9.0 * v);       // size of the dimension's terms at 3 sigma
             cond2 += tau * tau;
+            // what a point of this component adds to the accumulator in this dimension, on average (log2 units)
+            ramp += 0.5 * w * (m * m - v - (double)kap[d] / (s * s));
             mx = fmax(mx, fmax(fabs(a), fabs(b)));
         }
         ab_s[d] = a;
         ab_s[Dpad + d] = b;
     }
-    red[0][t] = mx; red[1][t] = csum; red[2][t] = cond2;
+    red[0][t] = mx; red[1][t] = csum; red[2][t] = cond2; red[4][t] = ramp;
     __syncthreads();
     for (int o = 128; o > 0; o >>= 1) {
         if (t < o) {
             red[0][t] = fmax(red[0][t], red[0][t + o]);
             red[1][t] += red[1][t + o];
             red[2][t] += red[2][t + o];
+            red[4][t] += red[4][t + o];
         }
         __syncthreads();
     }
@@ -814,15 +839,25 @@ __global__ void __launch_bounds__(256) wide_prepare_kernel(int D, int Dpad, int 
             const float pk = pi[k];
             if (pk > 0.f) c = 1.4426950408889634074 * (log((double)pk) - 0.5 * red[1][0]) - red[3][0];
         }
-        // error estimate of the approximate log2 z: operand rounding at 2^-22 of every term, terms of independent sign
-        const double est = 4.0 * 2.384185791015625e-07 * sqrt(red[2][0]);
+        // Error estimate of the approximate log2 z of the pairs that matter (points of the component itself).
+        // (i) operand rounding at 2^-22 of every term, terms of independent sign.  (ii) The tensor core truncates its fp32
+        // accumulator at each of the Dpad / 8 steps of the main product, by half an ulp (2^-24 relative) on average and
+        // always toward zero: with the accumulator climbing to A = |mean drift of the component| + 2 standard deviations
+        // of the walk (each dimension adds (log2 e / 2)(z^2 - 1), standard deviation 1.02), that is about
+        // (Dpad / 16) 2^-23 A.  The drift is what kap_d cannot remove: kap_d centres the mixture's average component,
+        // a component whose sum_d (mu'^2 - var) / var is far from that average keeps the difference.
+        const double est_round = 4.0 * 2.384185791015625e-07 * sqrt(red[2][0]);
+        const double est_trunc = (double)Dpad / 16.0 * 1.1920928955078125e-07 * (fabs(red[4][0]) + 2.04 * sqrt((double)D));
+        const double est = fmax(est_round, est_trunc);
         // A component that holds few points (pi_k N below a threshold) is evaluated exactly as well: its parameters are
         // averages over few responsibilities, which for a component far from most of its points are formed from large
         // accumulators (|log2 z - c_k| in the thousands) whose truncation error nothing averages out.
         float margin = 0.f;
         if (k < K && pi[k] > 0.f && (!(est <= (double)cond_limit) || pi[k] < min_weight)) {
-            // (flagged for its weight alone: a tiny positive mark, which the list kernel uses to keep the two kinds apart)
-            margin = !(est <= (double)cond_limit) ? (float)fmin(fmax(8.0 * est, 1e-10), 1e30) : 1e-30f;
+            // (Two kinds, kept apart by the list kernel.  Flagged by the rounding estimate: narrow in some or all dimensions,
+            // hopeless for most points -- the mark is its error bound.  Flagged for its drift or its weight alone: broad --
+            // a tiny positive mark.)
+            margin = !(est_round <= (double)cond_limit) ? (float)fmin(fmax(8.0 * est_round, 1e-10), 1e30) : 1e-30f;
             if (!(margin > 0.f)) margin = 1e30f;
             atomicOr(flags, 1);
             atomicAdd(flags + 4, 1);

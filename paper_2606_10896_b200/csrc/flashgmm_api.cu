@@ -274,9 +274,11 @@ bool auto_is_tensor(int D, int K) { return tc_supports(D, K) && K >= 64 && D >= 
 // AUTO also uses the tensor-core assignment for the larger K that only the assignment kernels take: planes are needed then
 // (and for D > 128 the two-sweep tensor path, which needs its own planes)
 bool auto_wants_planes(int D, int K) { return (tc_assign_supports(D, K) && K >= 64 && D >= 8) || (wide_supports(D, K) && K >= 64); }
-// Points per component from which AUTO takes the tensor path for D > 128: its logits carry an error of about 1e-4 in the
-// log2 domain (fp32 accumulators of magnitude ~100), which the averaging over a component's points must absorb.
-constexpr int64_t WIDE_AUTO_MIN_POINTS_PER_COMPONENT = 32;
+// Points per component from which AUTO takes the tensor path for D > 128.  Its logits carry an error of a few 1e-4 in the
+// log2 domain (fp32 accumulators of magnitude ~100, truncated at every step), which the averaging over a component's
+// points must absorb; components expected to hold fewer than wide_min_points (64) points are evaluated exactly, and
+// with fewer than about twice that per component on average most components would be.
+constexpr int64_t WIDE_AUTO_MIN_POINTS_PER_COMPONENT = 128;
 
 int ensure_scratch(gmm_ctx* ctx, int D, int K) {
     const bool planes = (tc_assign_supports(D, K) || wide_supports(D, K)) &&

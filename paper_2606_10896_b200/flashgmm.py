@@ -76,6 +76,7 @@ EXPORTS = {
     "gmm_kernel_time": (ctypes.c_int, [ctypes.c_void_p, ctypes.POINTER(ctypes.c_double),
                                        ctypes.POINTER(ctypes.c_int64)]),
     "gmm_reset_counters": (ctypes.c_int, [ctypes.c_void_p]),
+    "gmm_probe_rates": (ctypes.c_int, [ctypes.c_int, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]),
     "gmm_strerror": (ctypes.c_char_p, [ctypes.c_int]),
     "gmm_last_error": (ctypes.c_char_p, [ctypes.c_void_p]),
     "gmm_version": (ctypes.c_char_p, []),
@@ -110,6 +111,15 @@ def tensor_path_supports(D: int, K: int) -> bool:
 
 def gmm_auto_path(D: int, K: int) -> int:
     return int(lib.gmm_auto_path(int(D), int(K)))
+
+
+def gmm_probe_rates(device: int = 0):
+    """(fp32 FMA flop/s, ex2 results/s) measured on the device by two short micro-benchmarks."""
+    a, b = ctypes.c_double(0.0), ctypes.c_double(0.0)
+    rc = lib.gmm_probe_rates(int(device), ctypes.byref(a), ctypes.byref(b))
+    if rc != GMM_OK:
+        raise GmmError(rc, "gmm_probe_rates failed")
+    return a.value, b.value
 
 
 def gmm_scratch_bytes(D: int, K: int) -> int:

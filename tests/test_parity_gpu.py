@@ -764,38 +764,105 @@ def test_config4_full_size_conservation_additivity_and_subsample(fg, ctx):
     assert_stats_close(len(rows), data_scale(Xsub), got[:3], ref[:3], "config 4 subsample")
 
 
-def test_config5_shape_step_and_topm_on_subsample(fg, ctx):
-    """The IVF coarse-quantizer shape (D = 768, K = 4096, unit-norm vectors): one EM step and top-4 assignment on
-    1M device-generated points (AUTO path = the FP32 kernels: the shape is outside the tensor path), conservation at
-    that N, and the oracle on a seeded 20K-row subsample for both the step and the top-4 output."""
+def _config5_subsample_check(fg, ctx, X, spec, pi0, mu0, var0, idx, resp, p1, m1, v1):
+    """Oracle on a seeded 20K-row subsample: one EM step from the initial parameters (the GPU re-runs it on the same
+    rows; with 5 points per component AUTO takes the FP32 kernels there) and the top-4 rows of the full-size assignment."""
+    rows = synth.subsample_rows(spec.N, 20_000, spec.seed)
+    rows_d = torch.as_tensor(rows, device=DEV)
+    Xsub_d = X[rows_d].contiguous()
+    Xsub = Xsub_d.cpu().numpy()
+    ref = orc.em_step(Xsub, pi0, mu0, var0)
+    ctx.gmm_set_path(fg.GMM_PATH_AUTO)
+    got = _gpu_step(ctx, Xsub_d, pi0, mu0, var0)
+    assert abs(got[3] - ref[3]) <= 1e-5 * abs(ref[3])
+    assert_stats_close(len(rows), data_scale(Xsub), got[:3], ref[:3], "config 5 subsample")
+    _check_topm(Xsub, p1, m1, v1, 4, idx[rows_d].cpu().numpy(), resp[rows_d].cpu().numpy(), "config 5 top-4 subsample")
+
+
+def _params_from(ctx, N, stats, var_floor, pi, mu, var):
+    pi_d, mu_d, var_d = _t(pi), _t(mu), _t(var)
+    ctx.gmm_finalize(N, _t(stats[0], torch.float64), _t(stats[1], torch.float64), _t(stats[2], torch.float64), var_floor,
+                     pi_d, mu_d, var_d)
+    return pi_d.cpu().numpy(), mu_d.cpu().numpy(), var_d.cpu().numpy()
+
+
+def test_config5_shape_tensor_path_against_fp32_path_and_oracle_subsample(fg, ctx):
+    """The IVF coarse-quantizer shape (D = 768, K = 4096, unit-norm vectors) on 1M device-generated points, the launch
+    configuration the benchmark times (AUTO = the two-sweep tensor path).  No oracle run of this size is affordable, so:
+    conservation laws at that N; the tensor path against the FP32 kernels (which have no approximation to tune, and are
+    themselves checked against the oracle on the subsample below) over the SAME 1M rows at the ordinary tolerances, at
+    the initial parameters and at the parameters five EM iterations later (sharp posteriors, a thousand components
+    collapsed onto single points, hundreds that hold a few dozen points); the oracle on a seeded 20K-row subsample for
+    the step and the top-4 output."""
     spec = synth.CONFIGS[5].with_n(1_000_000)
+    X = synth.sample_device(spec, DEV)
+    pi0, mu0, var0 = synth.init_params(X, spec)
+    N = spec.N
+    s = float(np.sqrt(synth.global_variance(X[:200_000]).mean()))
+    col1, col2 = _column_sums(X)
+    pi, mu, var = pi0, mu0, var0
+    for stage in ("initial parameters", "after 5 iterations"):
+        ctx.gmm_set_path(fg.GMM_PATH_AUTO)
+        t_ = _gpu_step(ctx, X, pi, mu, var)
+        assert ctx.gmm_last_path() == fg.GMM_PATH_TENSOR, stage
+        assert abs(t_[0].sum() - N) <= 1e-5 * N
+        np.testing.assert_allclose(t_[2].sum(0), col2, rtol=1e-4)
+        np.testing.assert_allclose(t_[1].sum(0), col1, rtol=1e-4, atol=1e-4 * N * 0.04)
+        ctx.gmm_set_path(fg.GMM_PATH_FP32)
+        f_ = _gpu_step(ctx, X, pi, mu, var)
+        what = f"config 5 shape, 1M rows, tensor vs FP32 path, {stage}"
+        assert abs(t_[3] - f_[3]) <= 1e-5 * abs(f_[3]), what
+        assert_stats_close(N, s, t_[:3], f_[:3], what)
+        assert_params_close(N, s, _params_from(ctx, N, t_, spec.var_floor, pi, mu, var),
+                            _params_from(ctx, N, f_, spec.var_floor, pi, mu, var), f_[0], what)
+        if stage == "initial parameters":
+            ctx.gmm_set_path(fg.GMM_PATH_AUTO)
+            pi_d, mu_d, var_d = _t(pi0), _t(mu0), _t(var0)
+            ctx.gmm_fit(X, pi_d, mu_d, var_d, 5, spec.var_floor)
+            pi, mu, var = pi_d.cpu().numpy(), mu_d.cpu().numpy(), var_d.cpu().numpy()
+    assert ctx.gmm_last_exact_count() == 0            # (the last step ran on the FP32 path)
+    # parameters after one update from the initial ones for the top-m check, as config 5 prescribes after its fit
+    ctx.gmm_set_path(fg.GMM_PATH_AUTO)
+    st = _gpu_step(ctx, X, pi0, mu0, var0)
+    p1, m1, v1 = _params_from(ctx, N, st, spec.var_floor, pi0, mu0, var0)
+    idx, resp = ctx.gmm_assign_topm(X, _t(p1), _t(m1), _t(v1), 4)
+    torch.cuda.synchronize()
+    _config5_subsample_check(fg, ctx, X, spec, pi0, mu0, var0, idx, resp, p1, m1, v1)
+
+
+def test_config5_full_size_fit_and_assignment(fg, ctx):
+    """Config 5 as stated: N = 10M (30.7 GB of X), 20 EM iterations (gmm_fit, AUTO path), then gmm_assign_topm with m = 4
+    over all N; conservation at full N, a non-decreasing log-likelihood trace, device memory in use independent of N,
+    the oracle on a seeded 20K-row subsample for one step and for the top-4 output."""
+    spec = synth.CONFIGS[5]
+    free_b, _ = torch.cuda.mem_get_info()
+    if free_b < 40e9:
+        pytest.skip("needs 40 GB of free device memory")
     X = synth.sample_device(spec, DEV)
     pi0, mu0, var0 = synth.init_params(X, spec)
     N = spec.N
     col1, col2 = _column_sums(X)
     ctx.gmm_set_path(fg.GMM_PATH_AUTO)
-    Nk, S1, S2, L = _gpu_step(ctx, X, pi0, mu0, var0)
-    assert ctx.gmm_last_path() == fg.GMM_PATH_FP32
+    pi_d, mu_d, var_d = _t(pi0), _t(mu0), _t(var0)
+    ctx.gmm_em_step(X[:300_000], pi_d, mu_d, var_d)               # allocates the scratch
+    torch.cuda.synchronize()
+    free_small = torch.cuda.mem_get_info()[0]
+    trace, done = ctx.gmm_fit(X, pi_d, mu_d, var_d, spec.iters, spec.var_floor)
+    assert done == spec.iters == 20 and ctx.gmm_last_path() == fg.GMM_PATH_TENSOR
+    assert torch.cuda.mem_get_info()[0] == free_small, "device memory in use changed with N"
+    assert np.all(np.isfinite(trace))
+    # (variances pinned at the floor and frozen empty components may break the monotone growth by a hair)
+    assert (np.diff(trace) >= -1e-7 * np.abs(trace[1:])).all(), trace
+    Nk, S1, S2, L = _gpu_step(ctx, X, pi_d.cpu().numpy(), mu_d.cpu().numpy(), var_d.cpu().numpy())
     assert abs(Nk.sum() - N) <= 1e-5 * N
     np.testing.assert_allclose(S2.sum(0), col2, rtol=1e-4)
     np.testing.assert_allclose(S1.sum(0), col1, rtol=1e-4, atol=1e-4 * N * 0.04)
-    # parameters after one update (sharper responsibilities) for the top-m check
-    pi_d, mu_d, var_d = _t(pi0), _t(mu0), _t(var0)
-    ctx.gmm_finalize(N, _t(Nk, torch.float64), _t(S1, torch.float64), _t(S2, torch.float64), spec.var_floor, pi_d, mu_d,
-                     var_d)
+    assert L >= trace[-1] - 1e-7 * abs(L)
     idx, resp = ctx.gmm_assign_topm(X, pi_d, mu_d, var_d, 4)
     torch.cuda.synchronize()
-    rows = synth.subsample_rows(N, 20_000, spec.seed)
-    rows_d = torch.as_tensor(rows, device=DEV)
-    Xsub_d = X[rows_d].contiguous()
-    Xsub = Xsub_d.cpu().numpy()
-    ref = orc.em_step(Xsub, pi0, mu0, var0)
-    got = _gpu_step(ctx, Xsub_d, pi0, mu0, var0)
-    assert abs(got[3] - ref[3]) <= 1e-5 * abs(ref[3])
-    assert_stats_close(len(rows), data_scale(Xsub), got[:3], ref[:3], "config 5 subsample")
-    p1, m1, v1 = pi_d.cpu().numpy(), mu_d.cpu().numpy(), var_d.cpu().numpy()
-    _check_topm(Xsub, p1, m1, v1, 4, idx[rows_d].cpu().numpy(), resp[rows_d].cpu().numpy(),
-                "config 5 top-4 subsample")
+    assert int(idx.min()) >= 0 and int(idx.max()) < spec.K
+    _config5_subsample_check(fg, ctx, X, spec, pi0, mu0, var0, idx, resp, pi_d.cpu().numpy(), mu_d.cpu().numpy(),
+                             var_d.cpu().numpy())
 
 
 def test_isotropic_update_and_fit_match_the_papers_model(fg, ctx):

@@ -1,0 +1,172 @@
+"""GPU parity of the tensor-core path for wide data (128 < D <= 1024: the two sweeps of Algorithm 1 on tcgen05) against
+the float64 CPU oracle, through the C ABI.  Tolerances: tests/parity_util.py (the same as for every other path).
+
+What the path does with the components it cannot treat through the expanded quadratic form (collapsed ones, and ones
+that hold few points) is part of what is tested: they are evaluated exactly by the FP32 kernels as a packed
+sub-mixture, and gmm_last_exact_count reports how many there were.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import gmm_oracle as orc
+from paper_2606_10896_b200 import synth
+from tests.parity_util import assert_params_close, assert_stats_close, data_scale
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module")
+def fg():
+    from paper_2606_10896_b200 import flashgmm
+
+    return flashgmm
+
+
+@pytest.fixture()
+def ctx(fg):
+    c = fg.Context(0)
+    yield c
+    c.close()
+
+
+def _t(a, dtype=torch.float32):
+    return torch.as_tensor(np.ascontiguousarray(a), dtype=dtype, device=DEV).contiguous()
+
+
+def _clustered(rng, N, D, K, sep=0.3, spread=0.3):
+    """K clusters of about N / K points each (weights between 0.5 and 1.5 of the mean), parameters near the truth.  Centres
+    and noise are of the same size per dimension (sum_d mu^2 / var about D, as for unit-norm embeddings); in hundreds of
+    dimensions the clusters are still tens of standard deviations apart."""
+    centres = (rng.normal(size=(K, D)) * sep).astype(np.float32)
+    w = rng.uniform(0.5, 1.5, K)
+    w /= w.sum()
+    z = rng.choice(K, size=N, p=w)
+    sig = rng.uniform(0.7, 1.3, size=(K, D)) * spread
+    X = (centres[z] + rng.normal(size=(N, D)) * sig[z]).astype(np.float32)
+    mu = (centres + 0.05 * spread * rng.normal(size=(K, D))).astype(np.float32)
+    var = (sig ** 2 * rng.uniform(0.8, 1.25, size=(K, D))).astype(np.float32)
+    pi = w.astype(np.float32)
+    return X, pi, mu, var
+
+
+def _step_and_check(fg, ctx, X, pi, mu, var, what, var_floor=1e-6):
+    N = len(X)
+    s = data_scale(X)
+    ref = orc.em_step(X, pi, mu, var)
+    pr, mr, vr, _, _, _ = orc.em_iteration(X, pi, mu, var, var_floor=var_floor)
+    Nk, S1, S2, L = ctx.gmm_em_step(_t(X), _t(pi), _t(mu), _t(var))
+    got = (Nk.cpu().numpy(), S1.cpu().numpy(), S2.cpu().numpy())
+    assert abs(L - ref[3]) <= 1e-5 * abs(ref[3]), f"{what}: loglik {L} vs {ref[3]}"
+    assert abs(got[0].sum() - N) <= 1e-5 * N, f"{what}: sum N_k = {got[0].sum()}"
+    assert_stats_close(N, s, got, ref[:3], what)
+    pi_d, mu_d, var_d = _t(pi), _t(mu), _t(var)
+    ctx.gmm_finalize(N, Nk, S1, S2, var_floor, pi_d, mu_d, var_d)
+    assert_params_close(N, s, (pi_d.cpu().numpy(), mu_d.cpu().numpy(), var_d.cpu().numpy()), (pr, mr, vr), ref[0], what)
+    return got
+
+
+@pytest.mark.parametrize("N,D,K", [(20_000, 200, 130), (16_384 + 77, 768, 128), (30_000, 1024, 64), (25_000, 129, 70),
+                                   (40_000, 768, 256), (300, 256, 1)])
+def test_wide_tensor_path_one_step_against_oracle(fg, ctx, N, D, K):
+    """Ragged last slice of dimensions (200 = 128 + 72, 129), the largest D, a ragged last slice of components (130, 70),
+    tiles and batches with a ragged tail, one component."""
+    X, pi, mu, var = _clustered(np.random.default_rng(N + D + K), N, D, K)
+    assert fg.tensor_path_supports(D, K)
+    ctx.gmm_set_path(fg.GMM_PATH_TENSOR)
+    _step_and_check(fg, ctx, X, pi, mu, var, f"wide tensor N={N} D={D} K={K}")
+    assert ctx.gmm_last_path() == fg.GMM_PATH_TENSOR
+
+
+def test_wide_path_over_several_pieces_and_bit_identical_runs(fg, monkeypatch):
+    """Pieces of 1024 points (instead of 2^17): planes, log Z buffer and partial blocks are reused piece after piece; two
+    calls give the same bits."""
+    monkeypatch.setenv("GMM_WIDE_PIECE", "1024")
+    X, pi, mu, var = _clustered(np.random.default_rng(3), 5000, 384, 40)
+    with fg.Context(0) as c:
+        c.gmm_set_path(fg.GMM_PATH_TENSOR)
+        a = _step_and_check(fg, c, X, pi, mu, var, "five pieces")
+        Nk, S1, S2, L = c.gmm_em_step(_t(X), _t(pi), _t(mu), _t(var))
+        for u, v in zip(a, (Nk, S1, S2)):
+            assert np.array_equal(u, v.cpu().numpy())
+
+
+def test_wide_path_with_collapsed_and_low_weight_components(fg, ctx):
+    """Components collapsed onto a data point at the variance floor (the expanded form cannot represent them), components
+    narrow in a few dimensions only, and components of tiny weight: all are evaluated exactly, the rest on the tensor
+    cores, and the two must agree on the normaliser."""
+    rng = np.random.default_rng(17)
+    N, D, K = 30_000, 320, 96
+    X, pi, mu, var = _clustered(rng, N, D, K)
+    for j in range(6):                       # collapsed onto a point
+        mu[j] = X[100 + j]
+        var[j] = 1e-6
+    var[6:10, ::5] = 1e-5                    # narrow in every fifth dimension
+    pi[10:14] = 3e-4                         # about nine points' worth of weight each
+    pi = (pi / pi.sum()).astype(np.float32)
+    ctx.gmm_set_path(fg.GMM_PATH_TENSOR)
+    _step_and_check(fg, ctx, X, pi, mu, var, "collapsed / narrow / light components")
+    assert ctx.gmm_last_path() == fg.GMM_PATH_TENSOR
+    assert 10 <= ctx.gmm_last_exact_count() <= 20
+    # zero weights: no NaN, N_k = 0 there
+    pi2 = pi.copy()
+    pi2[20:30] = 0
+    pi2 = (pi2 / pi2.sum()).astype(np.float32)
+    got = _step_and_check(fg, ctx, X, pi2, mu, var, "zero weights")
+    assert np.all(got[0][20:30] == 0)
+
+
+def test_wide_auto_path_rule(fg, ctx):
+    """AUTO takes the tensor path for D > 128 from 128 points per component on (and K >= 64), the FP32 kernels below; a
+    parameter set in which more than half of the components need exact evaluation runs on the FP32 kernels too."""
+    rng = np.random.default_rng(5)
+    D, K = 256, 64
+    assert fg.gmm_auto_path(D, K) == fg.GMM_PATH_TENSOR and fg.gmm_auto_path(D, 32) == fg.GMM_PATH_FP32
+    X, pi, mu, var = _clustered(rng, 200 * K, D, K)
+    ctx.gmm_set_path(fg.GMM_PATH_AUTO)
+    ctx.gmm_em_step(_t(X), _t(pi), _t(mu), _t(var))
+    assert ctx.gmm_last_path() == fg.GMM_PATH_TENSOR
+    ctx.gmm_em_step(_t(X[:100 * K]), _t(pi), _t(mu), _t(var))
+    assert ctx.gmm_last_path() == fg.GMM_PATH_FP32
+    v2 = var.copy()
+    v2[:40] = 1e-6
+    ctx.gmm_em_step(_t(X), _t(pi), _t(mu), _t(v2))
+    assert ctx.gmm_last_path() == fg.GMM_PATH_FP32 and ctx.gmm_last_exact_count() == 0
+
+
+def test_wide_free_running_fit_matches_the_oracle_trace(fg, ctx):
+    rng = np.random.default_rng(9)
+    N, D, K = 20_000, 256, 64
+    X, pi, mu, var = _clustered(rng, N, D, K)
+    mu0 = X[rng.choice(N, K, replace=False)].copy()
+    var0 = np.tile(X.astype(np.float64).var(0).astype(np.float32), (K, 1))
+    pi0 = np.full(K, 1 / K, np.float32)
+    ref = orc.fit(X, pi0, mu0, var0, 10, var_floor=1e-6)
+    ctx.gmm_set_path(fg.GMM_PATH_TENSOR)
+    pi_d, mu_d, var_d = _t(pi0), _t(mu0), _t(var0)
+    trace, done = ctx.gmm_fit(_t(X), pi_d, mu_d, var_d, 10, 1e-6)
+    assert done == 10 and ctx.gmm_last_path() == fg.GMM_PATH_TENSOR
+    np.testing.assert_allclose(trace, ref["trace"], rtol=1e-4)
+    s = data_scale(X)
+    Nk = orc.em_step(X, ref["pi"], ref["mu"], ref["var"])[0]
+    assert np.abs(mu_d.cpu().numpy() - ref["mu"])[Nk >= 1].max() <= 1e-3 * s
+
+
+def test_wide_path_reports_non_finite_data(fg, ctx):
+    X, pi, mu, var = _clustered(np.random.default_rng(2), 3000, 200, 16)
+    X[77, 150] = np.nan
+    ctx.gmm_set_path(fg.GMM_PATH_TENSOR)
+    with pytest.raises(fg.GmmError) as e:
+        ctx.gmm_em_step(_t(X), _t(pi), _t(mu), _t(var))
+    assert e.value.code == fg.GMM_ENUMERIC
+    X[77, 150] = 0.0
+    ctx.gmm_em_step(_t(X), _t(pi), _t(mu), _t(var))
+
+
+def test_wide_data_far_from_the_origin(fg, ctx):
+    X, pi, mu, var = _clustered(np.random.default_rng(4), 12_000, 256, 48)
+    X = (X + 200.0).astype(np.float32)
+    mu = (mu + 200.0).astype(np.float32)
+    ctx.gmm_set_path(fg.GMM_PATH_TENSOR)
+    _step_and_check(fg, ctx, X, pi, mu, var, "wide, 200 units from the origin")

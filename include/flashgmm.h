@@ -230,7 +230,11 @@ int gmm_fisher_vectors(gmm_ctx* ctx, const float* X, int64_t N, const int64_t* o
  *   Always the FP32 path.  Results equal gmm_em_step's up to float32 summation order (the per-CTA partials are
  *   grouped differently), i.e. well inside the tolerances of the parity tests; they are still deterministic.
  *   The first call on each device looks up the array's device address (cudaGetSymbolAddress): make that first call
- *   before starting any stream capture.
+ *   before starting any stream capture.  The CUDA runtime also loads a kernel's code into the device the first time
+ *   that kernel is launched, which may allocate and synchronise inside the driver: a caller that must not allocate
+ *   from some point on makes one warm-up call per device and per kernel variant before that point -- the variants
+ *   are D <= 128 (float logits) and D > 128 (float64 logits, another M-step kernel).  The looked-up address is cached
+ *   per device for the life of the process; it does not survive cudaDeviceReset.
  *   Every call on a device shares the one array and the array keeps the previous call's contents; the function
  *   clears what it accumulates into, but two calls that overlap on the same GPU (different streams or threads)
  *   race on it -- serialise them.  Synchronises the stream before returning. */

@@ -4,8 +4,10 @@
 // a memory-budgeted service whose device heap is owned by another allocator, a plugin invoked between a framework's
 // own allocations where a driver allocation would synchronise the device, or a real-time loop that forbids any call
 // that can block on the driver's allocator.  For them this file keeps ALL scratch of the FP32 kernel chain in one
-// file-scope device array that is part of the loaded module: nothing is allocated or freed, here or in any routine
-// this entry point calls.
+// file-scope device array that is part of the loaded module: this file and the launch routines it calls make no
+// allocation call.  (What the CUDA runtime itself does on the FIRST launch of a kernel -- loading its code into the
+// device -- is outside this library's control: a warm-up call per device and per kernel variant, D <= 128 and
+// D > 128, puts that behind the caller.  The cached device address of the array does not survive cudaDeviceReset.)
 #include "internal.cuh"
 
 #include <cmath>

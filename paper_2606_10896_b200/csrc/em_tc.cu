@@ -1136,8 +1136,18 @@ __global__ void __launch_bounds__(128) tc_prepare_kernel(int D, int K, const flo
     // interleaved column order: k-step ks = d / 8 holds [x(8 dims) | x^2(8 dims)]
     const int cx = 16 * (d >> 3) + (d & 7), cq = cx + 8;
     hi_s[cx] = ah; hi_s[cq] = bh; lo_s[cx] = al; lo_s[cq] = bl;
-    // what the contraction adds through the shifted squares: t * (b_hi + b_lo) * kap, summed over d, is taken out of c_k
-    red_k[d] = live ? t * ((double)__half2float(bh) + (double)__half2float(bl)) * (double)kap[d] : 0.0;
+    // what the contraction adds through the shifted squares: t * (b_hi + b_lo) * kap, summed over d, is taken out of c_k.
+    // So is the effect of the coefficients' own rounding (a, b are kept to 22 bits of the row's largest entry: an error
+    // that is the same for every point, so nothing averages it out) AT THE COMPONENT'S MEAN: with ra, rb the residuals of
+    // the split, the contraction misses t (ra u + rb (u^2 + kap)); its value at u = s (mu - g) goes into c_k, and what is
+    // left is proportional to a point's distance from the mean, i.e. smaller by the component's |mu - g| / sigma.
+    {
+        const double bq = (double)__half2float(bh) + (double)__half2float(bl);
+        const double ra = as - ((double)__half2float(ah) + (double)__half2float(al)), rb = bs - bq;
+        double um = 0.0;
+        if (live) um = ((double)mu[(size_t)k * D + d] - (double)gd[d]) * (double)sd[d];
+        red_k[d] = live ? t * (bq * (double)kap[d] - (ra * um + rb * (um * um + (double)kap[d]))) : 0.0;
+    }
     __syncthreads();
     for (int o = 64; o > 0; o >>= 1) {
         if (d < o) red_k[d] += red_k[d + o];

@@ -823,8 +823,14 @@ __global__ void __launch_bounds__(256) wide_prepare_kernel(int D, int Dpad, int 
         const __half al = __double2half(as - (double)__half2float(ah)), bl = __double2half(bs - (double)__half2float(bh));
         const int cx = 16 * (d >> 3) + (d & 7);          // k-step interleaved column order, slices of 128 dimensions in sequence
         rh[cx] = ah; rh[cx + 8] = bh; rl[cx] = al; rl[cx + 8] = bl;
-        // what the contraction adds through the shifted squares is taken out of c_k
-        ksum += tt * ((double)__half2float(bh) + (double)__half2float(bl)) * (double)kap[d];
+        // what the contraction adds through the shifted squares is taken out of c_k; so is what the rounding of the
+        // coefficients (22 bits of the row's largest entry: the same error for every point) makes it miss at the
+        // component's own mean u = s (mu - g), which leaves an error proportional to a point's distance from that mean
+        const double bq = (double)__half2float(bh) + (double)__half2float(bl);
+        const double ra = as - ((double)__half2float(ah) + (double)__half2float(al)), rb = bs - bq;
+        double um = 0.0;
+        if (k < K && d < D) um = ((double)mu[(size_t)k * D + d] - (double)gd[d]) * (double)sd[d];
+        ksum += tt * (bq * (double)kap[d] - (ra * um + rb * (um * um + (double)kap[d])));
     }
     __syncthreads();
     red[3][t] = ksum;

@@ -31,8 +31,8 @@ def assert_params_close(N, s, got, ref, Nk_ref, what=""):
 
 
 def assert_stats_close(N, s, got, ref, what=""):
-    """Statistics compared on the scale the parameter tolerances imply: N_k to 1e-5 N; S1 to 1e-4 s max(N_k, 1);
-    S2 to 1e-4 s^2 max(N_k, 1), each plus a small share (1e-5 / 3e-5) of its own size.
+    """Statistics compared on the scale the parameter tolerances imply: N_k to 1e-5 N; S1 / N_k to 1e-4 s; S2 / N_k to
+    1e-4 s^2, each plus a small share (1e-5 / 3e-5) of its own size.
 
     Both sides are first moved to the data's centre c_d = sum_k S1_kd / sum_k N_k (S1' = S1 - c N_k,
     S2' = S2 - 2 c S1 + c^2 N_k, in float64): the parameters that follow from the statistics do not depend on where the
@@ -48,10 +48,14 @@ def assert_stats_close(N, s, got, ref, what=""):
 
     S1_g, S2_g = centred(Nk_g, S1_g, S2_g)
     S1_r, S2_r = centred(Nk_r, S1_r, S2_r)
-    w = np.maximum(Nk_r, 1.0)[:, None]
-    e1 = (np.abs(S1_g - S1_r) / w - 1e-5 * np.abs(S1_r) / w).max()
+    # Each side's sums are divided by its OWN N_k (at least 1): what is compared is the weighted mean and the weighted
+    # second moment a component implies.  A difference of 1e-6 in a component's total weight N_k scales all three of
+    # its statistics alike, moves pi_k by 1e-6 pi_k and mu_k, var_k not at all; divided by the other side's N_k it would
+    # show up multiplied by the component's distance from the centre squared.  (N_k itself is compared above.)
+    wg, wr = np.maximum(Nk_g, 1.0)[:, None], np.maximum(Nk_r, 1.0)[:, None]
+    e1 = (np.abs(S1_g / wg - S1_r / wr) - 1e-5 * np.abs(S1_r) / wr).max()
     assert e1 <= 1e-4 * s, f"{what}: S1/N_k off by {e1:.3e} > {1e-4 * s:.3e}"
-    e2 = (np.abs(S2_g - S2_r) / w - 3e-5 * (S2_r / w)).max()
+    e2 = (np.abs(S2_g / wg - S2_r / wr) - 3e-5 * (S2_r / wr)).max()
     assert e2 <= 1e-4 * s * s, f"{what}: S2/N_k off by {e2:.3e} > {1e-4 * s * s:.3e}"
 
 

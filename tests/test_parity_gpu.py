@@ -263,7 +263,9 @@ def test_forced_tensor_path_on_small_mixtures(fg, ctx, N, D, K):
 def test_auto_path_choice(fg, ctx):
     assert fg.gmm_auto_path(128, 1024) == fg.GMM_PATH_TENSOR
     assert fg.gmm_auto_path(16, 8) == fg.GMM_PATH_FP32
-    assert fg.gmm_auto_path(768, 4096) == fg.GMM_PATH_FP32 and not fg.tensor_path_supports(768, 4096)
+    # D > 128: the two-sweep tensor path (up to D = 1024), for which AUTO also looks at the points per component
+    assert fg.gmm_auto_path(768, 4096) == fg.GMM_PATH_TENSOR and fg.tensor_path_supports(768, 4096)
+    assert fg.gmm_auto_path(1025, 64) == fg.GMM_PATH_FP32 and not fg.tensor_path_supports(1025, 64)
     assert fg.gmm_auto_path(128, 4096) == fg.GMM_PATH_TENSOR and fg.gmm_auto_path(128, 4097) == fg.GMM_PATH_FP32
     X = _t(np.random.default_rng(0).normal(size=(500, 16)).astype(np.float32))
     pi, mu, var = _t(np.full(8, 1 / 8)), _t(np.random.default_rng(1).normal(size=(8, 16))), _t(np.ones((8, 16)))
@@ -692,6 +694,32 @@ def test_config3_full_size_conservation_and_subsample(fg, ctx):
     _full_size_topm_check(fg, ctx, X, spec, pi0, mu0, var0, "config 3, all rows, sampled")
 
 
+def test_config3_full_oracle_step_after_five_iterations(fg, ctx):
+    """Where the tensor path's accuracy knob is loose it must be checked against the oracle itself: the limit above which a
+    component's logits are recomputed exactly grows with sqrt(N / K) (4.7e-3 here against 1e-3 on a 50K-row subsample),
+    and after a few iterations from the data-row initialisation some components have collapsed onto points and others
+    are narrow in a few dimensions.  So: five EM iterations on the GPU (AUTO path), then ONE float64 oracle step over
+    all 1M rows at those parameters, compared per component at the ordinary tolerances."""
+    spec = synth.CONFIGS[3]
+    X = synth.sample_device(spec, DEV)
+    pi0, mu0, var0 = synth.init_params(X, spec)
+    N = spec.N
+    ctx.gmm_set_path(fg.GMM_PATH_AUTO)
+    pi_d, mu_d, var_d = _t(pi0), _t(mu0), _t(var0)
+    ctx.gmm_fit(X, pi_d, mu_d, var_d, 5, spec.var_floor)
+    p5, m5, v5 = pi_d.cpu().numpy(), mu_d.cpu().numpy(), var_d.cpu().numpy()
+    Xh = X.cpu().numpy()
+    s = data_scale(Xh[:200_000])
+    Nk_r, S1_r, S2_r, L_r = orc.em_step(Xh, p5, m5, v5)
+    pr, mr, vr = orc.finalize_moments(N, Nk_r, S1_r, S2_r, spec.var_floor, m5.astype(np.float64), v5.astype(np.float64))
+    got = _gpu_step(ctx, X, p5, m5, v5)
+    assert ctx.gmm_last_path() == fg.GMM_PATH_TENSOR and ctx.gmm_last_exact_count() > 0
+    what = "config 3, all 1M rows, after 5 iterations, AUTO path vs oracle"
+    assert abs(got[3] - L_r) <= 1e-5 * abs(L_r), what
+    assert_stats_close(N, s, got[:3], (Nk_r, S1_r, S2_r), what)
+    assert_params_close(N, s, _params_from(ctx, N, got, spec.var_floor, p5, m5, v5), (pr, mr, vr), Nk_r, what)
+
+
 def _full_size_topm_check(fg, ctx, X, spec, pi0, mu0, var0, what, n_rows=3000):
     """Top-4 assignment over ALL rows of X, as bench.py --assign-m 4 launches it, under the parameters one EM iteration
     gives; a seeded sample of rows is compared with the oracle's assignment of those rows one by one."""
@@ -753,6 +781,25 @@ def test_config4_full_size_conservation_additivity_and_subsample(fg, ctx):
     np.testing.assert_allclose(a[2] + b[2], S2, rtol=2e-5, atol=1e-5 * N / spec.K)
     assert abs((a[3] + b[3]) - L) <= 1e-9 * abs(L)
     _full_size_topm_check(fg, ctx, X, spec, pi0, mu0, var0, "config 4, all rows, sampled")
+    # The regime the benchmark times: parameters after five iterations (collapsed and narrow components; the exact
+    # recomputation protocol active with the limit of N = 100M, 4.7e-2, fifty times that of the subsample check below).
+    # No oracle run of this size is affordable; the FP32 kernels (no approximation to tune; themselves checked against
+    # the oracle) take all 100M rows in six seconds, so the tensor path is compared with them over ALL rows at the
+    # ordinary tolerances.
+    ctx.gmm_set_path(fg.GMM_PATH_AUTO)
+    pi_d, mu_d, var_d = _t(pi0), _t(mu0), _t(var0)
+    ctx.gmm_fit(X, pi_d, mu_d, var_d, 5, spec.var_floor)
+    p5, m5, v5 = pi_d.cpu().numpy(), mu_d.cpu().numpy(), var_d.cpu().numpy()
+    t_ = _gpu_step(ctx, X, p5, m5, v5)
+    assert ctx.gmm_last_path() == fg.GMM_PATH_TENSOR and ctx.gmm_last_exact_count() > 0
+    ctx.gmm_set_path(fg.GMM_PATH_FP32)
+    f_ = _gpu_step(ctx, X, p5, m5, v5)
+    what = "config 4, all 100M rows, after 5 iterations, tensor vs FP32 path"
+    assert abs(t_[3] - f_[3]) <= 1e-5 * abs(f_[3]), what
+    assert_stats_close(N, s, t_[:3], f_[:3], what)
+    assert_params_close(N, s, _params_from(ctx, N, t_, spec.var_floor, p5, m5, v5),
+                        _params_from(ctx, N, f_, spec.var_floor, p5, m5, v5), f_[0], what)
+    ctx.gmm_set_path(fg.GMM_PATH_AUTO)
     # oracle on a seeded subsample, GPU re-run on the same rows
     rows = synth.subsample_rows(N, 50_000, spec.seed)
     Xsub_d = X[torch.as_tensor(rows, device=DEV)].contiguous()

@@ -462,7 +462,8 @@ template <bool EARLY>
 __global__ void __launch_bounds__(NTHREADS, 2)
 mstep_wide_kernel(const float* __restrict__ X, int64_t n, int D, int K, const float* __restrict__ mu,
                   const float* __restrict__ w2, const double* __restrict__ c2, const float* __restrict__ g,
-                  const double* __restrict__ logZ2, double* __restrict__ partials) {
+                  const double* __restrict__ logZ2, double* __restrict__ partials, const int* __restrict__ run_if) {
+    if (run_if && run_if[0] == 0) return;          // gated launch: see lse_kernel
     extern __shared__ __align__(16) unsigned char smem_raw[];
     TileSmem& sm = *reinterpret_cast<TileSmem*>(smem_raw);
     float* r_all = reinterpret_cast<float*>(smem_raw + sizeof(TileSmem));   // [WT][TP][LDR]
@@ -709,12 +710,12 @@ static inline bool fp32_high_precision(int D) { return D > 128; }
 
 cudaError_t launch_lse_fp32(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu,
                             const float* w2, const double* c2d, const float* g, double* logZ2, double* llpart,
-                            const double* lower2) {
+                            const double* lower2, const int* run_if) {
     const unsigned blocks = (unsigned)((n + TP - 1) / TP);
     if (fp32_high_precision(D))
-        lse_kernel<0, double><<<blocks, NTHREADS, sizeof(TileSmem), s>>>(X, n, D, K, mu, w2, c2d, g, logZ2, llpart, 0, nullptr, nullptr, nullptr, nullptr, nullptr, lower2);
+        lse_kernel<0, double><<<blocks, NTHREADS, sizeof(TileSmem), s>>>(X, n, D, K, mu, w2, c2d, g, logZ2, llpart, 0, nullptr, nullptr, run_if, nullptr, nullptr, lower2);
     else
-        lse_kernel<0, float><<<blocks, NTHREADS, sizeof(TileSmem), s>>>(X, n, D, K, mu, w2, c2d, g, logZ2, llpart, 0, nullptr, nullptr, nullptr, nullptr, nullptr);
+        lse_kernel<0, float><<<blocks, NTHREADS, sizeof(TileSmem), s>>>(X, n, D, K, mu, w2, c2d, g, logZ2, llpart, 0, nullptr, nullptr, run_if, nullptr, nullptr);
     return cudaGetLastError();
 }
 
@@ -761,7 +762,7 @@ cudaError_t launch_topm_fp32(cudaStream_t s, const float* X, int64_t n, int D, i
 
 cudaError_t launch_mstep_fp32(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu,
                               const float* w2, const double* c2d, const float* g, const double* logZ2, float* partials,
-                              const Fp32Plan& plan, bool early) {
+                              const Fp32Plan& plan, bool early, const int* run_if) {
     if (plan.wide) {
         cudaError_t e = early ? cudaFuncSetAttribute(mstep_wide_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)MSTEP_WIDE_SMEM)
                               : cudaFuncSetAttribute(mstep_wide_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)MSTEP_WIDE_SMEM);
@@ -770,8 +771,8 @@ cudaError_t launch_mstep_fp32(cudaStream_t s, const float* X, int64_t n, int D, 
         e = cudaMemsetAsync(partials, 0, bytes, s);          // the kernel accumulates into its partials
         if (e != cudaSuccess) return e;
         dim3 wgrid(plan.comp_blocks, plan.splits, 1);
-        if (early) mstep_wide_kernel<true><<<wgrid, NTHREADS, MSTEP_WIDE_SMEM, s>>>(X, n, D, K, mu, w2, c2d, g, logZ2, reinterpret_cast<double*>(partials));
-        else mstep_wide_kernel<false><<<wgrid, NTHREADS, MSTEP_WIDE_SMEM, s>>>(X, n, D, K, mu, w2, c2d, g, logZ2, reinterpret_cast<double*>(partials));
+        if (early) mstep_wide_kernel<true><<<wgrid, NTHREADS, MSTEP_WIDE_SMEM, s>>>(X, n, D, K, mu, w2, c2d, g, logZ2, reinterpret_cast<double*>(partials), run_if);
+        else mstep_wide_kernel<false><<<wgrid, NTHREADS, MSTEP_WIDE_SMEM, s>>>(X, n, D, K, mu, w2, c2d, g, logZ2, reinterpret_cast<double*>(partials), run_if);
         return cudaGetLastError();
     }
     dim3 grid(plan.comp_blocks, plan.splits, plan.d_chunks);

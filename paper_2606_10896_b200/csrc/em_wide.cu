@@ -62,6 +62,15 @@ struct LseParams {
     double* llpart;
     float4* top;         // [n] per point: its two largest approximate log2 z (relative to c_ref) and their components
     int* status;
+    // screening of the listed (ill-conditioned) components, all NULL / 0 when there are none
+    const float2* scr;   // [NC * 128] (c_k - c_ref + allowance, allowance per unit of |x - g|^2); -inf for unlisted components
+    const int* scr_mask; // [NC * 4] nonzero where a chunk of 32 components holds a listed one
+    const int* slot_of;  // [NC * 128]
+    const float* n2;     // [n]
+    unsigned* cand;      // [n][cand_words]
+    int cand_words;
+    int scr_group;       // first group of 256 columns that holds listed components (they hold nothing else from there on)
+    int* ctl;
 };
 
 __global__ void __launch_bounds__(WT_THREADS, 1)
@@ -76,6 +85,7 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
     float2* merge_s = reinterpret_cast<float2*>(smem + L_MERGE);
     double* ll_s = reinterpret_cast<double*>(smem + L_MERGE);      // after the last tile
     __shared__ float4 top_s[128];
+    __shared__ float xm_s[256];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int64_t ntiles = (p.n + WIDE_TILE - 1) / WIDE_TILE;
@@ -116,10 +126,19 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
         for (int64_t i = 0; i < ntl; ++i) {
             const int64_t row = (blockIdx.x + i * gridDim.x) * WIDE_TILE + pt;
             float m_run = -1e30f, s_run = 0.f;               // finite start: blocks of -inf logits must not make NaN
+            const float nrm = (p.scr != nullptr && row < p.n) ? __ldg(p.n2 + row) : 0.f;
+            float thr_base = -1e30f;
+            int nhit = 0;
             float t1 = -CUDART_INF_F, t2 = -CUDART_INF_F;    // the two largest logits of this thread's chunks, and where
             int i1 = -1, i2 = -1;
             for (int g = 0; g < NG; ++g) {
                 const int nch = (NC - 2 * g < 2) ? (NC - 2 * g) : 2;
+                const bool screening = p.scr != nullptr && g >= p.scr_group;
+                if (screening && g == p.scr_group) {          // the two warpgroups' running maxima, merged once per tile
+                    xm_s[grp * 128 + pt] = m_run;
+                    named_bar_sync(3, 256);
+                    thr_base = fmaxf(m_run, xm_s[(grp ^ 1) * 128 + pt]);
+                }
                 const bool got = bar_wait(BAR(LB_LFULL), uses & 1u, abort_flag, p.status, false);
                 const bool ok = __all_sync(0xffffffffu, got);
                 fence_after();
@@ -136,6 +155,31 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
                             tmem_wait_ld();
                             const int col0 = (2 * g + c) * 128 + sub * 32;
                             const float4* tc4 = reinterpret_cast<const float4*>(p.tkck + col0);
+                            if (screening) {
+                                // Columns of listed components (they take no part in the sums): their approximate values,
+                                // raised by what they can be wrong by, tell which pairs can matter at all.  The point's
+                                // maximum over the evaluated components is final by now.  (!(a < b): a NaN passes.)
+                                if (__ldg(p.scr_mask + (col0 >> 5)) != 0 && row < p.n) {
+                                    const float thr = thr_base - 40.f;
+                                    const float4* sc4 = reinterpret_cast<const float4*>(p.scr + col0);
+#pragma unroll
+                                    for (int j = 0; j < 32; j += 2) {
+                                        const float4 q = __ldg(tc4 + (j >> 1));
+                                        const float4 sq = __ldg(sc4 + (j >> 1));
+                                        const float u0 = fmaf(__uint_as_float(v[j]) + __uint_as_float(vc[j]), q.x, fmaf(sq.y, nrm, sq.x));
+                                        const float u1 = fmaf(__uint_as_float(v[j + 1]) + __uint_as_float(vc[j + 1]), q.z, fmaf(sq.w, nrm, sq.z));
+                                        if (!(u0 < thr) && sq.x > -CUDART_INF_F) {
+                                            const int sl = __ldg(p.slot_of + col0 + j);
+                                            if (sl >= 0) { atomicOr(p.cand + row * p.cand_words + (sl >> 5), 1u << (sl & 31)); ++nhit; }
+                                        }
+                                        if (!(u1 < thr) && sq.z > -CUDART_INF_F) {
+                                            const int sl = __ldg(p.slot_of + col0 + j + 1);
+                                            if (sl >= 0) { atomicOr(p.cand + row * p.cand_words + (sl >> 5), 1u << (sl & 31)); ++nhit; }
+                                        }
+                                    }
+                                }
+                                continue;
+                            }
                             float l[32];
                             float bmax = -CUDART_INF_F;
 #pragma unroll
@@ -199,6 +243,7 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
                     ll_acc += lz;
                 }
             }
+            if (nhit > 0) atomicAdd(p.ctl, nhit);
             named_bar_sync(2, 256);                          // merge_s is rewritten by the next tile
         }
         if (grp == 0) ll_s[pt] = ll_acc;
@@ -771,43 +816,174 @@ __global__ void __launch_bounds__(128) wide_scale_kernel(int D, int K, const flo
     }
 }
 
-// One block per padded component: coefficient planes, t_k, c_k (float64), conditioning flag.
-__global__ void __launch_bounds__(256) wide_prepare_kernel(int D, int Dpad, int K, const float* __restrict__ pi,
+// One block per component: the error estimate of its approximate logits, and whether the tensor passes may take it.
+// Error estimate of the approximate log2 z of the pairs that matter (points of the component itself).
+// (i) operand rounding at 2^-22 of every term, terms of independent sign.  (ii) The tensor core truncates its fp32
+// accumulator at each of the Dpad / 8 steps of the main product, by half an ulp (2^-24 relative) on average and
+// always toward zero: with the accumulator climbing to A = |mean drift of the component| + 2 standard deviations
+// of the walk (each dimension adds (log2 e / 2)(z^2 - 1), standard deviation 1.02), that is about
+// (Dpad / 16) 2^-23 A.  The drift is what kap_d cannot remove: kap_d centres the mixture's average component,
+// a component whose sum_d (mu'^2 - var) / var is far from that average keeps the difference.
+// A component that holds few points (pi_k N below a threshold) is evaluated exactly as well: its parameters are
+// averages over few responsibilities, which for a component far from most of its points are formed from large
+// accumulators (|log2 z - c_k| in the thousands) whose truncation error nothing averages out.
+// Output: illb[k] > 0 for a flagged component (two kinds, kept apart by the list kernel.  Flagged by the rounding estimate:
+// narrow in some or all dimensions, hopeless for most points -- the mark is 8 x that estimate.  Flagged for its drift or its
+// weight alone: broad -- a tiny positive mark); scra[k], scrw[k]: what the approximate log2 z of ANY point can be wrong by
+// is at most scra + scrw |x - g|^2.  (Every term a u + b (u^2 + kap) is formed from operands kept to 2^-22 and added
+// into an accumulator that loses up to 2^-23 of its size at each of at most 128 steps, so the error is below 2^-15 times
+// the sum of the terms' sizes, and sum_d w (|mu' x'| + (x'^2 + |kap'|) / 2) <= sum_d w (mu'^2 + |kap'|) / 2 + max_d w |x'|^2.)
+__global__ void __launch_bounds__(256) wide_flag_kernel(int D, int Dpad, int K, const float* __restrict__ pi,
+                                                        const float* __restrict__ mu, const float* __restrict__ var,
+                                                        const float* __restrict__ sd, const float* __restrict__ kap,
+                                                        const float* __restrict__ gd, float* __restrict__ illb,
+                                                        float* __restrict__ scra, float* __restrict__ scrw,
+                                                        float cond_limit, float min_weight, int* __restrict__ flags) {
+    __shared__ double red[4][256];
+    const int k = blockIdx.x, t = threadIdx.x;
+    double cond2 = 0.0, ramp = 0.0, asum = 0.0, wmax = 0.0;
+    if (k < K)
+        for (int d = t; d < D; d += 256) {
+            const double v = (double)var[(size_t)k * D + d], m = (double)mu[(size_t)k * D + d] - (double)gd[d], s = (double)sd[d];
+            const double w = 1.4426950408889634074 / v;
+            const double kp = (double)kap[d] / (s * s);
+            const double tau = 0.5 * w * 3.0 * (m * m + 9.0 * v);       // size of the dimension's terms at 3 sigma
+            cond2 += tau * tau;
+            // what a point of this component adds to the accumulator in this dimension, on average (log2 units)
+            ramp += 0.5 * w * (m * m - v - kp);
+            asum += 0.5 * w * (m * m + fabs(kp));
+            wmax = fmax(wmax, w);
+        }
+    red[0][t] = cond2; red[1][t] = ramp; red[2][t] = asum; red[3][t] = wmax;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) {
+        if (t < o) {
+            red[0][t] += red[0][t + o];
+            red[1][t] += red[1][t + o];
+            red[2][t] += red[2][t + o];
+            red[3][t] = fmax(red[3][t], red[3][t + o]);
+        }
+        __syncthreads();
+    }
+    if (t == 0) {
+        const double est_round = 4.0 * 2.384185791015625e-07 * sqrt(red[0][0]);
+        const double est_trunc = (double)Dpad / 16.0 * 1.1920928955078125e-07 * (fabs(red[1][0]) + 2.04 * sqrt((double)D));
+        const double est = fmax(est_round, est_trunc);
+        float margin = 0.f;
+        if (k < K && pi[k] > 0.f && (!(est <= (double)cond_limit) || pi[k] < min_weight)) {
+            margin = !(est_round <= (double)cond_limit) ? (float)fmin(fmax(8.0 * est_round, 1e-10), 1e30) : 1e-30f;
+            if (!(margin > 0.f)) margin = 1e30f;
+            atomicOr(flags, 1);
+            atomicAdd(flags + 4, 1);
+        }
+        illb[k] = margin;
+        const double eps = 3.0517578125e-05;                 // 2^-15
+        const double a = 8.0 * est + eps * red[2][0] + 0.0625, w = eps * red[3][0];
+        scra[k] = (float)fmin(isfinite(a) ? a : 1e30, 1e30);
+        scrw[k] = (float)fmin(isfinite(w) ? w : 1e30, 1e30);
+    }
+}
+
+// Where each component sits in the tensor passes, and the list of the flagged ones.  One block of 1024 threads.
+// Positions [0, Kg): the components the tensor passes evaluate, in ascending order (flags[6] = Kg); [Kg, Kgp = the next
+// multiple of 256): empty; from Kgp on: the flagged components in the order of the list, which sweep 1 only screens (its
+// groups of 256 columns then hold either kind, never both, and every point's running maximum is final when the
+// screening starts).  comp_of[pos] = component or -1; slot_of[pos] = slot in the list or -1; scr_mask[pos / 32].
+// The list (at most WIDE_MAX_ILL slots; flags[2] = its length): first, in ascending order, the components flagged by
+// their error estimate (mostly collapsed onto a point), then, from the next multiple of 64 on (flags[5]; the gap is
+// filled with -1 = empty slots), those flagged for their drift or weight alone (broad): the FP32 kernels that evaluate the
+// list densely when the pairs are too many leave a tile of 64 collapsed components after its first chunk of dimensions.
+__global__ void __launch_bounds__(1024) wide_ill_list_kernel(int K, int rows, const float* __restrict__ illb, int* __restrict__ list,
+                                                             int* __restrict__ comp_of, int* __restrict__ slot_of,
+                                                             int* __restrict__ scr_mask, int* __restrict__ flags) {
+    __shared__ int wcount[32];
+    __shared__ int kgp_s;
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    for (int j = threadIdx.x; j < rows; j += 1024) { comp_of[j] = -1; slot_of[j] = -1; }
+    __syncthreads();
+    int done = 0;        // list slots used so far (kinds 0, 1) / positions used so far (kind 2 = the others)
+    int nflag = 0;       // flagged components placed so far
+    for (int kind = 2; kind >= 0; kind = (kind == 2 ? 0 : (kind == 0 ? 1 : -1))) {
+        if (kind == 0) done = 0;
+        for (int base = 0; base < K; base += 1024) {
+            const int k = base + threadIdx.x;
+            const float e = k < K ? illb[k] : -1.f;
+            const bool is = kind == 2 ? (e == 0.f) : (kind == 0 ? (e > 1e-20f) : (e > 0.f && e <= 1e-20f));
+            const unsigned b = __ballot_sync(0xffffffffu, is);
+            __syncthreads();
+            if (lane == 0) wcount[w] = __popc(b);
+            __syncthreads();
+            int before = 0, total = 0;
+            for (int j = 0; j < 32; ++j) {
+                if (j < w) before += wcount[j];
+                total += wcount[j];
+            }
+            const int rank = before + __popc(b & ((1u << lane) - 1u));
+            if (is) {
+                if (kind == 2) {
+                    comp_of[done + rank] = k;
+                } else if (done + rank < WIDE_MAX_ILL) {
+                    list[done + rank] = k;
+                    const int pos = kgp_s + nflag + rank;
+                    if (pos < rows) { comp_of[pos] = k; slot_of[pos] = done + rank; }
+                }
+            }
+            done += total;
+            if (kind != 2) nflag += total;
+        }
+        if (kind == 2) {
+            if (threadIdx.x == 0) { flags[6] = done; kgp_s = (done + 255) & ~255; }
+            __syncthreads();
+        }
+        if (kind == 0) {
+            const int padded = (done + 63) & ~63;
+            for (int j = done + threadIdx.x; j < padded && j < WIDE_MAX_ILL; j += 1024) list[j] = -1;
+            done = padded < WIDE_MAX_ILL ? padded : done;
+            if (threadIdx.x == 0) flags[5] = done;            // where the second kind starts
+            __syncthreads();
+        }
+    }
+    if (threadIdx.x == 0) flags[2] = done < WIDE_MAX_ILL ? done : WIDE_MAX_ILL;
+    __syncthreads();
+    for (int c = threadIdx.x; c < rows / 32; c += 1024) {
+        int any = 0;
+        for (int j = 0; j < 32; ++j) any |= (slot_of[32 * c + j] >= 0) ? 1 : 0;
+        scr_mask[c] = any;
+    }
+}
+
+// One block per position of the tensor passes: coefficient planes, t, c (float64) of the component that sits there
+// (zero planes and c = -inf for an empty position).
+__global__ void __launch_bounds__(256) wide_prepare_kernel(int D, int Dpad, const int* __restrict__ comp_of, const float* __restrict__ pi,
                                                            const float* __restrict__ mu, const float* __restrict__ var,
                                                            const float* __restrict__ sd, const float* __restrict__ kap,
                                                            const float* __restrict__ gd, __half* __restrict__ p_hi,
                                                            __half* __restrict__ p_lo, float* __restrict__ tk,
-                                                           double* __restrict__ ckd, float* __restrict__ illb,
-                                                           float cond_limit, float min_weight, int* __restrict__ flags) {
+                                                           double* __restrict__ ckd) {
     extern __shared__ double ab_s[];                     // [2][Dpad]: a, b of this component
-    __shared__ double red[5][256];
-    const int k = blockIdx.x, t = threadIdx.x;
-    double mx = 0.0, csum = 0.0, cond2 = 0.0, ramp = 0.0;
+    __shared__ double red[3][256];
+    const int pos = blockIdx.x, t = threadIdx.x;
+    const int k = comp_of[pos];
+    double mx = 0.0, csum = 0.0;
     for (int d = t; d < Dpad; d += 256) {
         double a = 0.0, b = 0.0;
-        if (k < K && d < D) {
+        if (k >= 0 && d < D) {
             const double v = (double)var[(size_t)k * D + d], m = (double)mu[(size_t)k * D + d] - (double)gd[d], s = (double)sd[d];
             const double w = 1.4426950408889634074 / v;
             a = w * m / s;
             b = -0.5 * w / (s * s);
             csum += m * m / v + log(6.283185307179586476925286766559 * v);
-            const double tau = 0.5 * w * 3.0 * (m * m + 9.0 * v);       // size of the dimension's terms at 3 sigma
-            cond2 += tau * tau;
-            // what a point of this component adds to the accumulator in this dimension, on average (log2 units)
-            ramp += 0.5 * w * (m * m - v - (double)kap[d] / (s * s));
             mx = fmax(mx, fmax(fabs(a), fabs(b)));
         }
         ab_s[d] = a;
         ab_s[Dpad + d] = b;
     }
-    red[0][t] = mx; red[1][t] = csum; red[2][t] = cond2; red[4][t] = ramp;
+    red[0][t] = mx; red[1][t] = csum;
     __syncthreads();
     for (int o = 128; o > 0; o >>= 1) {
         if (t < o) {
             red[0][t] = fmax(red[0][t], red[0][t + o]);
             red[1][t] += red[1][t + o];
-            red[2][t] += red[2][t + o];
-            red[4][t] += red[4][t + o];
         }
         __syncthreads();
     }
@@ -815,8 +991,8 @@ __global__ void __launch_bounds__(256) wide_prepare_kernel(int D, int Dpad, int 
     double tt = 1.0;
     if (mx > 0.0 && isfinite(mx)) tt = exp2(floor(log2(mx)) - 9.0);      // max |P / t| in [512, 1024)
     double ksum = 0.0;
-    __half* rh = p_hi + (size_t)k * 2 * Dpad;
-    __half* rl = p_lo + (size_t)k * 2 * Dpad;
+    __half* rh = p_hi + (size_t)pos * 2 * Dpad;
+    __half* rl = p_lo + (size_t)pos * 2 * Dpad;
     for (int d = t; d < Dpad; d += 256) {
         const double as = ab_s[d] / tt, bs = ab_s[Dpad + d] / tt;
         const __half ah = __double2half(as), bh = __double2half(bs);
@@ -829,59 +1005,39 @@ __global__ void __launch_bounds__(256) wide_prepare_kernel(int D, int Dpad, int 
         const double bq = (double)__half2float(bh) + (double)__half2float(bl);
         const double ra = as - ((double)__half2float(ah) + (double)__half2float(al)), rb = bs - bq;
         double um = 0.0;
-        if (k < K && d < D) um = ((double)mu[(size_t)k * D + d] - (double)gd[d]) * (double)sd[d];
+        if (k >= 0 && d < D) um = ((double)mu[(size_t)k * D + d] - (double)gd[d]) * (double)sd[d];
         ksum += tt * (bq * (double)kap[d] - (ra * um + rb * (um * um + (double)kap[d])));
     }
     __syncthreads();
-    red[3][t] = ksum;
+    red[2][t] = ksum;
     __syncthreads();
     for (int o = 128; o > 0; o >>= 1) {
-        if (t < o) red[3][t] += red[3][t + o];
+        if (t < o) red[2][t] += red[2][t + o];
         __syncthreads();
     }
     if (t == 0) {
         double c = -CUDART_INF;
-        if (k < K) {
+        if (k >= 0) {
             const float pk = pi[k];
-            if (pk > 0.f) c = 1.4426950408889634074 * (log((double)pk) - 0.5 * red[1][0]) - red[3][0];
+            if (pk > 0.f) c = 1.4426950408889634074 * (log((double)pk) - 0.5 * red[1][0]) - red[2][0];
         }
-        // Error estimate of the approximate log2 z of the pairs that matter (points of the component itself).
-        // (i) operand rounding at 2^-22 of every term, terms of independent sign.  (ii) The tensor core truncates its fp32
-        // accumulator at each of the Dpad / 8 steps of the main product, by half an ulp (2^-24 relative) on average and
-        // always toward zero: with the accumulator climbing to A = |mean drift of the component| + 2 standard deviations
-        // of the walk (each dimension adds (log2 e / 2)(z^2 - 1), standard deviation 1.02), that is about
-        // (Dpad / 16) 2^-23 A.  The drift is what kap_d cannot remove: kap_d centres the mixture's average component,
-        // a component whose sum_d (mu'^2 - var) / var is far from that average keeps the difference.
-        const double est_round = 4.0 * 2.384185791015625e-07 * sqrt(red[2][0]);
-        const double est_trunc = (double)Dpad / 16.0 * 1.1920928955078125e-07 * (fabs(red[4][0]) + 2.04 * sqrt((double)D));
-        const double est = fmax(est_round, est_trunc);
-        // A component that holds few points (pi_k N below a threshold) is evaluated exactly as well: its parameters are
-        // averages over few responsibilities, which for a component far from most of its points are formed from large
-        // accumulators (|log2 z - c_k| in the thousands) whose truncation error nothing averages out.
-        float margin = 0.f;
-        if (k < K && pi[k] > 0.f && (!(est <= (double)cond_limit) || pi[k] < min_weight)) {
-            // (Two kinds, kept apart by the list kernel.  Flagged by the rounding estimate: narrow in some or all dimensions,
-            // hopeless for most points -- the mark is its error bound.  Flagged for its drift or its weight alone: broad --
-            // a tiny positive mark.)
-            margin = !(est_round <= (double)cond_limit) ? (float)fmin(fmax(8.0 * est_round, 1e-10), 1e30) : 1e-30f;
-            if (!(margin > 0.f)) margin = 1e30f;
-            atomicOr(flags, 1);
-            atomicAdd(flags + 4, 1);
-        }
-        tk[k] = (float)tt;
-        ckd[k] = c;
-        illb[k] = margin;
+        tk[pos] = (float)tt;
+        ckd[pos] = c;
     }
 }
 
-// c_ref = the largest finite c_k; tkck[k] = (t_k, c_k - c_ref) in fp32 (-inf where the component takes no part).
-__global__ void __launch_bounds__(1024) wide_cref_kernel(int Kpad, const float* __restrict__ tk, const double* __restrict__ ckd,
-                                                         const float* __restrict__ illb, double* __restrict__ cref,
-                                                         float2* __restrict__ tkck) {
+// c_ref = the largest finite c among the positions the tensor passes evaluate; tkck[pos] = (t, c - c_ref) in fp32 (-inf
+// where the position takes no part); scr[pos] = (c - c_ref + scra, scrw) for a listed component, (-inf, 0) elsewhere.
+__global__ void __launch_bounds__(1024) wide_cref_kernel(int rows, const int* __restrict__ flags, const float* __restrict__ tk,
+                                                         const double* __restrict__ ckd, const int* __restrict__ comp_of,
+                                                         const int* __restrict__ slot_of, const float* __restrict__ scra,
+                                                         const float* __restrict__ scrw, double* __restrict__ cref,
+                                                         float2* __restrict__ tkck, float2* __restrict__ scr) {
     __shared__ double red[1024];
+    const int Kg = flags[6];
     double m = -CUDART_INF;
-    for (int k = threadIdx.x; k < Kpad; k += 1024)
-        if (!(illb[k] > 0.f) && isfinite(ckd[k])) m = fmax(m, ckd[k]);
+    for (int k = threadIdx.x; k < Kg; k += 1024)
+        if (isfinite(ckd[k])) m = fmax(m, ckd[k]);
     red[threadIdx.x] = m;
     __syncthreads();
     for (int o = 512; o > 0; o >>= 1) {
@@ -890,45 +1046,53 @@ __global__ void __launch_bounds__(1024) wide_cref_kernel(int Kpad, const float* 
     }
     const double r = isfinite(red[0]) ? red[0] : 0.0;
     if (threadIdx.x == 0) *cref = r;
-    for (int k = threadIdx.x; k < Kpad; k += 1024) {
-        const bool in = !(illb[k] > 0.f) && isfinite(ckd[k]);
+    for (int k = threadIdx.x; k < rows; k += 1024) {
+        const bool in = k < Kg && isfinite(ckd[k]);
         tkck[k] = make_float2(tk[k], in ? (float)(ckd[k] - r) : -CUDART_INF_F);
+        const int c = comp_of[k];
+        const bool listed = slot_of[k] >= 0 && c >= 0 && isfinite(ckd[k]);
+        scr[k] = listed ? make_float2((float)fmin(ckd[k] - r + (double)scra[c], 3e38), scrw[c]) : make_float2(-CUDART_INF_F, 0.f);
     }
 }
 
 // stats += sum over the R partial blocks of a component slice (fixed order, float64), undoing the responsibility scale,
 // the per-dimension scale and centre, and the column order; the partial blocks are left as they are (the caller clears them).
-__global__ void wide_reduce_kernel(int D, int K, int CL, int R, int pcols, const float* __restrict__ partial,
-                                   const float* __restrict__ sd, const float* __restrict__ kap, const float* __restrict__ gd,
-                                   double* __restrict__ Nk, double* __restrict__ S1, double* __restrict__ S2) {
-    const size_t KD = (size_t)K * D, per = (size_t)K + 2 * KD;
+__global__ void wide_reduce_kernel(int D, int Kg, int CL, int R, int pcols, const float* __restrict__ partial,
+                                   const int* __restrict__ comp_of, const float* __restrict__ sd, const float* __restrict__ kap,
+                                   const float* __restrict__ gd, double* __restrict__ Nk, double* __restrict__ S1,
+                                   double* __restrict__ S2) {
+    // Kg: the positions the sweep evaluated; position p holds component comp_of[p]
+    const size_t KD = (size_t)Kg * D, per = (size_t)Kg + 2 * KD;
     const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (e >= per) return;
     const double unscale = 1.0 / (double)TC_RSCALE;
-    auto column = [&](int col, int k) {
+    auto column = [&](int col, int pos) {
         double s = 0.0;
-        const int sl = k >> 7, kl = k & 127;
+        const int sl = pos >> 7, kl = pos & 127;
         for (int q = 0; q < R; ++q) s += (double)partial[((size_t)(q * CL + sl) * pcols + col) * 128 + kl];
         return s;
     };
-    if (e < (size_t)K) {
-        const int k = (int)e;
-        Nk[e] += (column(pcols - 2, k) + column(pcols - 1, k)) * unscale;
+    if (e < (size_t)Kg) {
+        const int pos = (int)e, k = comp_of[pos];
+        if (k >= 0) Nk[k] += (column(pcols - 2, pos) + column(pcols - 1, pos)) * unscale;
         return;
     }
-    const bool second = e >= K + KD;
-    const size_t j = second ? (e - K - KD) : (e - K);
-    const int k = (int)(j / D), d = (int)(j % D);
+    const bool second = e >= Kg + KD;
+    const size_t j = second ? (e - Kg - KD) : (e - Kg);
+    const int pos = (int)(j / D), d = (int)(j % D);
+    const int k = comp_of[pos];
+    if (k < 0) return;
+    const size_t o = (size_t)k * D + d;
     const int col = 16 * (d >> 3) + (d & 7);
     const double s_d = (double)sd[d], g = (double)gd[d];
-    const double nk_raw = column(pcols - 2, k) + column(pcols - 1, k);
+    const double nk_raw = column(pcols - 2, pos) + column(pcols - 1, pos);
     const double nk = nk_raw * unscale;
-    const double s1c = column(col, k) * unscale / s_d;
+    const double s1c = column(col, pos) * unscale / s_d;
     if (!second) {
-        S1[j] += s1c + g * nk;
+        S1[o] += s1c + g * nk;
     } else {
-        const double s2c = (column(col + 8, k) - (double)kap[d] * nk_raw) * unscale / (s_d * s_d);
-        S2[j] += s2c + 2.0 * g * s1c + g * g * nk;
+        const double s2c = (column(col + 8, pos) - (double)kap[d] * nk_raw) * unscale / (s_d * s_d);
+        S2[o] += s2c + 2.0 * g * s1c + g * g * nk;
     }
 }
 
@@ -942,8 +1106,8 @@ __global__ void wide_reduce_kernel(int D, int K, int CL, int R, int pcols, const
 __global__ void __launch_bounds__(256) wide_refine_kernel(const float* __restrict__ X, int64_t n, int D, int K,
                                                           const float* __restrict__ mu, const float* __restrict__ w2,
                                                           const double* __restrict__ c2d, const double* __restrict__ cref,
-                                                          const float4* __restrict__ top, const double* __restrict__ logz,
-                                                          double* __restrict__ logz_x) {
+                                                          const float4* __restrict__ top, const int* __restrict__ comp_of,
+                                                          const double* __restrict__ logz, double* __restrict__ logz_x) {
     const int64_t i = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (i >= n) return;
@@ -955,7 +1119,7 @@ __global__ void __launch_bounds__(256) wide_refine_kernel(const float* __restric
     double corr = 0.0;
 #pragma unroll
     for (int c = 0; c < 2; ++c) {
-        const int k = ak[c];
+        const int k = (ak[c] >= 0) ? __ldg(comp_of + ak[c]) : -1;     // the sweep reports positions
         if (k < 0 || k >= K) continue;                       // warp-uniform
         const float* mr = mu + (size_t)k * D;
         const float* wr = w2 + (size_t)k * D;
@@ -983,47 +1147,7 @@ __global__ void __launch_bounds__(256) wide_refine_kernel(const float* __restric
     }
 }
 
-// ---- ill-conditioned components: evaluated exactly by the FP32 kernels as a sub-mixture -------------------------------
-// List of the flagged components (illb > 0), at most WIDE_MAX_ILL; one block of 1024 threads.  First, in ascending order,
-// those flagged by their error estimate (mostly components collapsed onto a point: hopeless for every other point, which
-// the FP32 tile routine notices after its first chunk of dimensions -- but only if ALL 64 components of its tile are of
-// that kind), then those flagged for their small weight alone (broad: they need the full evaluation).
-__global__ void __launch_bounds__(1024) wide_ill_list_kernel(int Kpad, const float* __restrict__ illb, int* __restrict__ list,
-                                                             int* __restrict__ flags) {
-    __shared__ int wcount[32];
-    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    int done = 0;
-    for (int kind = 0; kind < 2; ++kind) {
-        for (int base = 0; base < Kpad; base += 1024) {
-            const int k = base + threadIdx.x;
-            const float e = k < Kpad ? illb[k] : 0.f;
-            const bool is = kind == 0 ? (e > 1e-20f) : (e > 0.f && e <= 1e-20f);
-            const unsigned b = __ballot_sync(0xffffffffu, is);
-            __syncthreads();
-            if (lane == 0) wcount[w] = __popc(b);
-            __syncthreads();
-            int before = 0, total = 0;
-            for (int j = 0; j < 32; ++j) {
-                if (j < w) before += wcount[j];
-                total += wcount[j];
-            }
-            const int pos = done + before + __popc(b & ((1u << lane) - 1u));
-            if (is && pos < WIDE_MAX_ILL) list[pos] = k;
-            done += total;
-        }
-        if (kind == 0) {
-            // pad the first kind to a whole tile of 64 components with repeats of... nothing: the second kind simply starts
-            // at the next multiple of 64 (the gap is filled with component -1 = an empty slot)
-            const int padded = (done + 63) & ~63;
-            for (int j = done + threadIdx.x; j < padded && j < WIDE_MAX_ILL; j += 1024) list[j] = -1;
-            done = padded < WIDE_MAX_ILL ? padded : done;
-            if (threadIdx.x == 0) flags[5] = done;            // where the second kind starts
-            __syncthreads();
-        }
-    }
-    if (threadIdx.x == 0) flags[2] = done < WIDE_MAX_ILL ? done : WIDE_MAX_ILL;
-}
-
+// ---- ill-conditioned components: evaluated exactly, as a packed sub-mixture -------------------------------------------
 // The listed components' rows of mu, w2 and their constants, packed: the sub-mixture the FP32 kernels evaluate.
 __global__ void wide_ill_gather_kernel(int D, int n_ill, const int* __restrict__ list, const float* __restrict__ mu,
                                        const float* __restrict__ w2, const double* __restrict__ c2d, float* __restrict__ mu_c,
@@ -1067,6 +1191,201 @@ __global__ void __launch_bounds__(256) wide_merge_ll_kernel(int64_t n, double* _
         __syncthreads();
     }
     if (threadIdx.x == 0) llpart[blockIdx.x] += red[0] * 0.69314718055994530942;
+}
+
+// ---- the listed components evaluated pair by pair ---------------------------------------------------------------------
+// Sweep 1 marks the (point, listed component) pairs that can matter; at the paper's IVF sizes those are a few thousand
+// of the 10^8 pairs of a piece (a component collapsed onto a point matters for that point only), so evaluating them one
+// by one costs nothing next to the dense evaluation of the whole sub-mixture by the FP32 kernels, which stays as the
+// route for parameter sets in which the marked pairs are many (ctl[1]).
+
+// |x_i - g|^2 of the piece's points: one warp per point, fixed order.
+__global__ void __launch_bounds__(256) wide_norm_kernel(const float* __restrict__ X, int64_t n, int D, const float* __restrict__ gd,
+                                                        float* __restrict__ n2) {
+    const int64_t i = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (i >= n) return;
+    const float* xr = X + i * D;
+    float s = 0.f;
+    for (int d = lane; d < D; d += 32) {
+        const float t = __ldg(xr + d) - __ldg(gd + d);
+        s = fmaf(t, t, s);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) n2[i] = (s <= 3e38f) ? s : 3e38f;          // (a NaN or an infinity in X is reported by the transform kernel)
+}
+
+__global__ void wide_cand_gate_kernel(int* __restrict__ ctl, long long max_pairs) {
+    const int dense = ((long long)ctl[0] > max_pairs) ? 1 : 0;
+    ctl[1] = dense;
+    ctl[2] = 1 - dense;
+}
+
+// Per-step totals for diagnostics: flags[1] += pairs marked, flags[3] += pairs kept, flags[7] += 1 for a piece that went
+// through the dense kernels (saturating).
+__global__ void wide_cand_count_kernel(const int* __restrict__ ctl, int* __restrict__ flags) {
+    auto add = [](int a, int b) { const long long t = (long long)a + (long long)b; return t > 2147483647LL ? 2147483647 : (int)t; };
+    flags[1] = add(flags[1], ctl[0]);
+    flags[3] = add(flags[3], ctl[1] ? 0 : ctl[3]);
+    flags[7] = add(flags[7], ctl[1] ? 1 : 0);
+}
+
+// Exact log2 z of one pair by a whole warp: direct differences in fp32, a lane sums 4 dimensions of each 128 in fp32 and
+// adds the chunk sums in float64 (the arithmetic of the FP32 kernels and of wide_refine_kernel), fixed butterfly: every
+// lane returns the same bits.  The quadratic form only grows: once c - q (tracked in fp32, with a margin of 1) falls below
+// `stop` the rest cannot matter and -inf is returned.
+__device__ __forceinline__ double wide_pair_log2z(const float* __restrict__ xr, const float* __restrict__ mr,
+                                                  const float* __restrict__ wr, double c, int D, int lane, double stop) {
+    double q = 0.0;
+    float run = 0.f;
+    const float room = (stop > -CUDART_INF) ? (float)fmin(fmax(c - stop + 1.0, -3e38), 3e38) : CUDART_INF_F;
+    for (int d0 = 0; d0 < D; d0 += 128) {
+        float part = 0.f;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int d = d0 + lane + 32 * j;
+            if (d < D) {
+                const float diff = __ldg(xr + d) - __ldg(mr + d);
+                part = fmaf(diff * diff, __ldg(wr + d), part);
+            }
+        }
+        q += (double)part;
+        float tot = part;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, o);
+        run += tot;
+        if (run > room) return -CUDART_INF;                  // warp-uniform: tot is the same in every lane
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
+    return c - q;
+}
+
+// One warp per point: its marked pairs in ascending slot order; those within 2^-40 of the point's log2 Z over the
+// evaluated components (logz) are kept: log-sum-exp into out[i], bit (slot, i) of the transposed map.
+__global__ void __launch_bounds__(256) wide_cand_lse_kernel(const float* __restrict__ X, int64_t n, int D, int words,
+                                                            const unsigned* __restrict__ cand, unsigned* __restrict__ candT,
+                                                            const float* __restrict__ mu_c, const float* __restrict__ w2_c,
+                                                            const double* __restrict__ c2d_c, const double* __restrict__ logz,
+                                                            double* __restrict__ out, int* __restrict__ ctl) {
+    if (ctl[1] != 0) return;
+    const int64_t i = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (i >= n) return;
+    const unsigned b0 = (lane < words) ? cand[i * words + lane] : 0u;
+    const unsigned b1 = (lane + 32 < words) ? cand[i * words + 32 + lane] : 0u;
+    if (!__any_sync(0xffffffffu, (b0 | b1) != 0u)) {
+        if (lane == 0) out[i] = -CUDART_INF;
+        return;
+    }
+    const double lim = logz[i] - 40.0;
+    const float* xr = X + i * D;
+    double m = -CUDART_INF, ssum = 0.0;
+    int kept = 0;
+    for (int wi = 0; wi < words; ++wi) {
+        unsigned word = __shfl_sync(0xffffffffu, wi < 32 ? b0 : b1, wi & 31);
+        while (word) {
+            const int b = __ffs(word) - 1;
+            word &= word - 1;
+            const int slot = wi * 32 + b;
+            const double c = __ldg(c2d_c + slot);
+            const double l = wide_pair_log2z(xr, mu_c + (size_t)slot * D, w2_c + (size_t)slot * D, c, D, lane, lim);
+            if (l >= lim && l > -CUDART_INF) {               // warp-uniform
+                if (l > m) { ssum = ssum * exp2(m - l) + 1.0; m = l; }
+                else ssum += exp2(l - m);
+                if (lane == 0) atomicOr(candT + (size_t)slot * WIDE_CANDT_WORDS + (i >> 5), 1u << (i & 31));
+                ++kept;
+            }
+        }
+    }
+    if (lane == 0) {
+        out[i] = kept ? m + log2(ssum) : -CUDART_INF;
+        if (kept) atomicAdd(ctl + 3, kept);
+    }
+}
+
+// One block per slot: the points marked for it, in ascending order, 2048 rows of the map at a time: r = 2^(exact log2 z
+// - log2 Z) by one warp per pair, then every thread adds r (x - g), r (x - g)^2 for its dimensions (float64, the order
+// fixed: same bits in every run).  The sums are shifted back to the origin and added to the slot's statistics.
+__global__ void __launch_bounds__(256) wide_cand_mstep_kernel(const float* __restrict__ X, int64_t n, int D, const int* __restrict__ list,
+                                                              const unsigned* __restrict__ candT, const float* __restrict__ mu_c,
+                                                              const float* __restrict__ w2_c, const double* __restrict__ c2d_c,
+                                                              const float* __restrict__ gd, const double* __restrict__ logz_x,
+                                                              double* __restrict__ Nk_c, double* __restrict__ S1_c,
+                                                              double* __restrict__ S2_c, const int* __restrict__ ctl) {
+    if (ctl[1] != 0) return;
+    const int slot = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (list[slot] < 0) return;
+    const unsigned* bits = candT + (size_t)slot * WIDE_CANDT_WORDS;
+    const int words = (int)((n + 31) >> 5);
+    unsigned any = 0u;
+    for (int w = tid; w < words; w += 256) any |= bits[w];
+    if (!__syncthreads_or(any != 0u)) return;
+    __shared__ int rows_s[2048];
+    __shared__ double r_s[2048];
+    __shared__ int wsum[2];
+    const double c = c2d_c[slot];
+    const float* mr = mu_c + (size_t)slot * D;
+    const float* wr = w2_c + (size_t)slot * D;
+    double s1[4] = {0.0, 0.0, 0.0, 0.0}, s2[4] = {0.0, 0.0, 0.0, 0.0}, nk = 0.0;
+    float gq[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) gq[q] = (tid + 256 * q < D) ? gd[tid + 256 * q] : 0.f;
+    for (int w0 = 0; w0 < words; w0 += 64) {
+        unsigned word = (tid < 64 && w0 + tid < words) ? bits[w0 + tid] : 0u;
+        const int cnt = __popc(word);
+        int incl = cnt;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        if (warp < 2 && lane == 31) wsum[warp] = incl;
+        __syncthreads();
+        const int total = wsum[0] + wsum[1];
+        if (tid < 64) {
+            int at = (warp == 1 ? wsum[0] : 0) + incl - cnt;
+            while (word) {
+                const int b = __ffs(word) - 1;
+                word &= word - 1;
+                rows_s[at++] = (w0 + tid) * 32 + b;
+            }
+        }
+        __syncthreads();
+        if (total == 0) continue;                            // block-uniform
+        for (int e = warp; e < total; e += 8) {
+            const int row = rows_s[e];
+            const double l = wide_pair_log2z(X + (size_t)row * D, mr, wr, c, D, lane, -CUDART_INF);
+            if (lane == 0) r_s[e] = exp2(l - logz_x[row]);
+        }
+        __syncthreads();
+        for (int e = 0; e < total; ++e) {
+            const double r = r_s[e];
+            const float* xr = X + (size_t)rows_s[e] * D;
+            nk += r;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int d = tid + 256 * q;
+                if (d < D) {
+                    const double xd = (double)(__ldg(xr + d) - gq[q]);
+                    s1[q] += r * xd;
+                    s2[q] += r * xd * xd;
+                }
+            }
+        }
+        __syncthreads();                                     // rows_s, r_s and wsum are rewritten by the next round
+    }
+    if (tid == 0) Nk_c[slot] += nk;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        const int d = tid + 256 * q;
+        if (d < D) {
+            const double g = (double)gq[q];
+            S1_c[(size_t)slot * D + d] += s1[q] + g * nk;
+            S2_c[(size_t)slot * D + d] += s2[q] + 2.0 * g * s1[q] + g * g * nk;
+        }
+    }
 }
 
 // The sub-mixture's statistics go to the rows of its components (which the tensor passes left at zero).
@@ -1121,6 +1440,7 @@ WidePlan wide_plan(int D, int K, int num_sms) {
     pl.Dpad = pl.n_slices * 128;
     pl.CL = (K + 127) / 128;
     pl.Kpad = pl.CL * 128;
+    pl.rows = pl.Kpad + 256;
     pl.R = num_sms / pl.CL;
     if (pl.R < 1) pl.R = 1;
     pl.pcols = 2 * pl.Dpad + 2;
@@ -1135,18 +1455,20 @@ cudaError_t launch_prepare_wide(cudaStream_t s, int D, int K, const float* pi, c
     wide_scale_kernel<<<pl.Dpad, 128, 0, s>>>(D, K, pi, mu, var, wb.sd, wb.kap, wb.gd);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    wide_prepare_kernel<<<pl.Kpad, 256, (size_t)2 * pl.Dpad * sizeof(double), s>>>(
-        D, pl.Dpad, K, pi, mu, var, wb.sd, wb.kap, wb.gd, reinterpret_cast<__half*>(wb.p_hi), reinterpret_cast<__half*>(wb.p_lo),
-        wb.tk, wb.ckd, wb.illb, cond_limit, min_weight, wb.flags);
+    wide_flag_kernel<<<K, 256, 0, s>>>(D, pl.Dpad, K, pi, mu, var, wb.sd, wb.kap, wb.gd, wb.illb, wb.scra, wb.scrw, cond_limit,
+                                       min_weight, wb.flags);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    wide_cref_kernel<<<1, 1024, 0, s>>>(pl.Kpad, wb.tk, wb.ckd, wb.illb, wb.cref, reinterpret_cast<float2*>(wb.tkck));
-    return cudaGetLastError();
-}
-
-cudaError_t launch_ill_list_wide(cudaStream_t s, int D, int K, const WideBuffers& wb) {
-    const WidePlan pl = wide_plan(D, K, 148);
-    wide_ill_list_kernel<<<1, 1024, 0, s>>>(pl.Kpad, wb.illb, wb.ill_list, wb.flags);
+    wide_ill_list_kernel<<<1, 1024, 0, s>>>(K, pl.rows, wb.illb, wb.ill_list, wb.comp_of, wb.slot_of, wb.scr_mask, wb.flags);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    wide_prepare_kernel<<<pl.rows, 256, (size_t)2 * pl.Dpad * sizeof(double), s>>>(
+        D, pl.Dpad, wb.comp_of, pi, mu, var, wb.sd, wb.kap, wb.gd, reinterpret_cast<__half*>(wb.p_hi),
+        reinterpret_cast<__half*>(wb.p_lo), wb.tk, wb.ckd);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    wide_cref_kernel<<<1, 1024, 0, s>>>(pl.rows, wb.flags, wb.tk, wb.ckd, wb.comp_of, wb.slot_of, wb.scra, wb.scrw, wb.cref,
+                                        reinterpret_cast<float2*>(wb.tkck), reinterpret_cast<float2*>(wb.scr));
     return cudaGetLastError();
 }
 
@@ -1158,7 +1480,8 @@ cudaError_t launch_ill_gather_wide(cudaStream_t s, int D, int n_ill, const WideB
 
 cudaError_t launch_refine_wide(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu, const float* w2,
                                const double* c2d, const WideBuffers& wb) {
-    wide_refine_kernel<<<(unsigned)((n + 7) / 8), 256, 0, s>>>(X, n, D, K, mu, w2, c2d, wb.cref, reinterpret_cast<const float4*>(wb.top), wb.logz, wb.logz_x);
+    wide_refine_kernel<<<(unsigned)((n + 7) / 8), 256, 0, s>>>(X, n, D, K, mu, w2, c2d, wb.cref, reinterpret_cast<const float4*>(wb.top),
+                                                               wb.comp_of, wb.logz, wb.logz_x);
     return cudaGetLastError();
 }
 
@@ -1175,6 +1498,46 @@ cudaError_t launch_ill_scatter_wide(cudaStream_t s, int D, int K, int n_ill, con
     return cudaGetLastError();
 }
 
+cudaError_t launch_norm_wide(cudaStream_t s, const float* X, int64_t n, int D, const WideBuffers& wb) {
+    wide_norm_kernel<<<(unsigned)((n + 7) / 8), 256, 0, s>>>(X, n, D, wb.gd, wb.n2);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_cand_clear_wide(cudaStream_t s, int64_t n, int n_slots, const WideBuffers& wb) {
+    const int words = (n_slots + 31) / 32;
+    cudaError_t e = cudaMemsetAsync(wb.ctl, 0, 8 * sizeof(int), s);
+    if (e == cudaSuccess) e = cudaMemsetAsync(wb.cand, 0, (size_t)n * words * sizeof(unsigned), s);
+    if (e == cudaSuccess) e = cudaMemsetAsync(wb.candT, 0, (size_t)n_slots * WIDE_CANDT_WORDS * sizeof(unsigned), s);
+    return e;
+}
+
+cudaError_t launch_cand_gate_wide(cudaStream_t s, const WideBuffers& wb, long long max_pairs) {
+    wide_cand_gate_kernel<<<1, 1, 0, s>>>(wb.ctl, max_pairs);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_cand_count_wide(cudaStream_t s, const WideBuffers& wb) {
+    wide_cand_count_kernel<<<1, 1, 0, s>>>(wb.ctl, wb.flags);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_cand_lse_wide(cudaStream_t s, const float* X, int64_t n, int D, int n_slots, const WideBuffers& wb,
+                                 double* logz_ill) {
+    const int words = (n_slots + 31) / 32;
+    wide_cand_lse_kernel<<<(unsigned)((n + 7) / 8), 256, 0, s>>>(X, n, D, words, wb.cand, wb.candT, wb.mu_c, wb.w2_c, wb.c2d_c, wb.logz,
+                                                                 logz_ill, wb.ctl);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_cand_mstep_wide(cudaStream_t s, const float* X, int64_t n, int D, int n_slots, const WideBuffers& wb) {
+    double* Nk_c = wb.stats_c;
+    double* S1_c = Nk_c + n_slots;
+    double* S2_c = S1_c + (size_t)n_slots * D;
+    wide_cand_mstep_kernel<<<(unsigned)n_slots, 256, 0, s>>>(X, n, D, wb.ill_list, wb.candT, wb.mu_c, wb.w2_c, wb.c2d_c, wb.gd,
+                                                             wb.logz_x, Nk_c, S1_c, S2_c, wb.ctl);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_transform_wide(cudaStream_t s, const float* X, int64_t n, int D, const WideBuffers& wb, int* status) {
     if (n < 1 || n > WIDE_PIECE) return cudaErrorInvalidValue;
     const WidePlan pl = wide_plan(D, 1, 148);
@@ -1186,8 +1549,9 @@ cudaError_t launch_transform_wide(cudaStream_t s, const float* X, int64_t n, int
     return cudaGetLastError();
 }
 
-cudaError_t launch_lse_wide(cudaStream_t s, int64_t n, int D, int K, const WideBuffers& wb, int num_sms, int* status) {
-    if (n < 1 || n > WIDE_PIECE) return cudaErrorInvalidValue;
+cudaError_t launch_lse_wide(cudaStream_t s, int64_t n, int D, int K, int Kg, int n_listed, int n_slots, const WideBuffers& wb,
+                            int num_sms, int* status) {
+    if (n < 1 || n > WIDE_PIECE || Kg < 1 || Kg > K) return cudaErrorInvalidValue;
     const WidePlan pl = wide_plan(D, K, num_sms);
     const int64_t rp = rows_padded_of(n);
     const int64_t pitch = (int64_t)pl.Dpad * 4;
@@ -1195,29 +1559,37 @@ cudaError_t launch_lse_wide(cudaStream_t s, int64_t n, int D, int K, const WideB
     CUtensorMap tm_yhi, tm_ylo, tm_phi, tm_plo;
     cudaError_t e = wide_make_map(&tm_yhi, wb.y_hi, rp, pitch, atoms, WIDE_TILE, 1);
     if (e == cudaSuccess) e = wide_make_map(&tm_ylo, wb.y_lo, rp, pitch, atoms, WIDE_TILE, 1);
-    if (e == cudaSuccess) e = wide_make_map(&tm_phi, wb.p_hi, pl.Kpad, pitch, atoms, 128, 1);
-    if (e == cudaSuccess) e = wide_make_map(&tm_plo, wb.p_lo, pl.Kpad, pitch, atoms, 128, 1);
+    if (e == cudaSuccess) e = wide_make_map(&tm_phi, wb.p_hi, pl.rows, pitch, atoms, 128, 1);
+    if (e == cudaSuccess) e = wide_make_map(&tm_plo, wb.p_lo, pl.rows, pitch, atoms, 128, 1);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(lse_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L_SMEM);
     if (e != cudaSuccess) return e;
+    const int Kgp = (Kg + 255) & ~255;                   // where the listed components start
+    const bool screen = n_listed > 0 && n_slots > 0;
+    const int cols = screen ? (Kgp + n_listed) : Kg;
+    if (cols > pl.rows) return cudaErrorInvalidValue;
     LseParams p;
-    p.n = n; p.NC = pl.CL; p.NZ = atoms;
+    p.n = n; p.NC = (cols + 127) / 128; p.NZ = atoms;
     p.tkck = reinterpret_cast<const float2*>(wb.tkck); p.cref = wb.cref; p.logz = wb.logz; p.llpart = nullptr; p.status = status;
     p.top = reinterpret_cast<float4*>(wb.top);
+    p.scr = screen ? reinterpret_cast<const float2*>(wb.scr) : nullptr;
+    p.scr_mask = wb.scr_mask; p.slot_of = wb.slot_of; p.n2 = wb.n2; p.cand = wb.cand;
+    p.cand_words = (n_slots + 31) / 32; p.scr_group = Kgp / 256; p.ctl = wb.ctl;
     const int64_t ntiles = (n + WIDE_TILE - 1) / WIDE_TILE;
     const unsigned grid = (unsigned)(ntiles < num_sms ? ntiles : num_sms);
     lse_wide_kernel<<<grid, WT_THREADS, L_SMEM, s>>>(p, tm_yhi, tm_ylo, tm_phi, tm_plo);
     return cudaGetLastError();
 }
 
-cudaError_t launch_em_wide(cudaStream_t s, int64_t n, int D, int K, const WideBuffers& wb, int num_sms, int* status) {
-    if (n < 1 || n > WIDE_PIECE) return cudaErrorInvalidValue;
-    const WidePlan pl = wide_plan(D, K, num_sms);
+cudaError_t launch_em_wide(cudaStream_t s, int64_t n, int D, int K, int Kg, const WideBuffers& wb, int num_sms, int* status) {
+    if (n < 1 || n > WIDE_PIECE || Kg < 1 || Kg > K) return cudaErrorInvalidValue;
+    const WidePlan pk = wide_plan(D, K, num_sms);
+    const WidePlan pl = wide_plan(D, Kg, num_sms);       // the sweep covers the evaluated positions only
     const int64_t rp = rows_padded_of(n);
     const int64_t pitch = (int64_t)pl.Dpad * 4;
     const int atoms = 4 * pl.n_slices;
     CUtensorMap tm_phi, tm_plo, tm_ye_hi, tm_ye_lo, tm_ym_hi, tm_ym_lo;
-    cudaError_t e = wide_make_map(&tm_phi, wb.p_hi, pl.Kpad, pitch, atoms, 128, 1);
-    if (e == cudaSuccess) e = wide_make_map(&tm_plo, wb.p_lo, pl.Kpad, pitch, atoms, 128, 1);
+    cudaError_t e = wide_make_map(&tm_phi, wb.p_hi, pk.rows, pitch, atoms, 128, 1);
+    if (e == cudaSuccess) e = wide_make_map(&tm_plo, wb.p_lo, pk.rows, pitch, atoms, 128, 1);
     if (e == cudaSuccess) e = wide_make_map(&tm_ye_hi, wb.y_hi, rp, pitch, atoms, WIDE_BATCH, 1);
     if (e == cudaSuccess) e = wide_make_map(&tm_ye_lo, wb.y_lo, rp, pitch, atoms, WIDE_BATCH, 1);
     if (e == cudaSuccess) e = wide_make_map(&tm_ym_hi, wb.y_hi, rp, pitch, atoms, 64, 2);
@@ -1231,11 +1603,13 @@ cudaError_t launch_em_wide(cudaStream_t s, int64_t n, int D, int K, const WideBu
     return cudaGetLastError();
 }
 
-cudaError_t launch_reduce_wide(cudaStream_t s, int D, int K, const WideBuffers& wb, int num_sms, double* Nk, double* S1,
+cudaError_t launch_reduce_wide(cudaStream_t s, int D, int K, int Kg, const WideBuffers& wb, int num_sms, double* Nk, double* S1,
                                double* S2) {
-    const WidePlan pl = wide_plan(D, K, num_sms);
-    const size_t per = (size_t)K + 2 * (size_t)K * D;
-    wide_reduce_kernel<<<(unsigned)((per + 255) / 256), 256, 0, s>>>(D, K, pl.CL, pl.R, pl.pcols, wb.partial, wb.sd, wb.kap, wb.gd, Nk, S1, S2);
+    if (Kg < 1 || Kg > K) return cudaErrorInvalidValue;
+    const WidePlan pl = wide_plan(D, Kg, num_sms);       // the plan of the sweep that wrote the partial blocks
+    const size_t per = (size_t)Kg + 2 * (size_t)Kg * D;
+    wide_reduce_kernel<<<(unsigned)((per + 255) / 256), 256, 0, s>>>(D, Kg, pl.CL, pl.R, pl.pcols, wb.partial, wb.comp_of, wb.sd,
+                                                                     wb.kap, wb.gd, Nk, S1, S2);
     return cudaGetLastError();
 }
 

@@ -14,12 +14,16 @@ constexpr int WIDE_BATCH = 256;              // points per batch of the second s
 constexpr int WIDE_TILE = 128;               // points per tile of the first sweep
 constexpr int WIDE_MAX_ILL = 2048;           // ill-conditioned components the FP32 kernels evaluate as a sub-mixture
 constexpr int WIDE_LL_BLOCKS = 64;           // per-block partial sums of the log-likelihood
+constexpr int WIDE_CAND_WORDS = WIDE_MAX_ILL / 32;          // 32-bit words of a point's row of the candidate bitmap
+constexpr int WIDE_CANDT_WORDS = (int)(WIDE_PIECE / 32);    // words of a slot's row of the transposed bitmap
 
 struct WidePlan {
     int n_slices;   // ceil(D / 128): slices of 128 dimensions = 256 columns of the planes
     int Dpad;       // n_slices * 128
     int CL;         // ceil(K / 128) component slices
     int Kpad;       // CL * 128
+    int rows;       // Kpad + 256: rows of the coefficient planes and of the per-position arrays (the listed components sit
+                    // behind the evaluated ones, from the next multiple of 256 on)
     int R;          // point ranges of the second sweep: its grid is CL * R CTAs
     int pcols;      // columns of a partial block: 2 * Dpad statistics columns + 2 columns of N_k
 };
@@ -28,14 +32,19 @@ struct WideBuffers {
     float* sd;      // [Dpad] power-of-two scale of a dimension
     float* kap;     // [Dpad] constant added to the squares
     float* gd;      // [Dpad] centre subtracted from points and means
-    unsigned char* p_hi;   // [Kpad][2 Dpad] fp16: high parts of the scaled coefficients, k-step interleaved columns
+    // Arrays "by position": the tensor passes see the components in the order comp_of gives (evaluated ones first).
+    unsigned char* p_hi;   // [rows][2 Dpad] fp16: high parts of the scaled coefficients, k-step interleaved columns
     unsigned char* p_lo;   // the low parts
-    float* tk;      // [Kpad] row scale t_k
-    float* tkck;    // [Kpad] pairs (t_k, c_k - c_ref); c = -inf for padded, zero-weight and ill-conditioned components
-    double* ckd;    // [Kpad] c_k in float64
-    double* cref;   // [1] reference constant: the largest finite c_k
-    float* illb;    // [Kpad] > 0 for an ill-conditioned component
-    int* flags;     // [8]: [0] any ill-conditioned component, [4] how many, [2] slots of the list, [5] slots of its first kind
+    float* tk;      // [rows] row scale t
+    float* tkck;    // [rows] pairs (t, c - c_ref); c = -inf for empty positions, zero-weight and listed components
+    double* ckd;    // [rows] c in float64
+    double* cref;   // [1] reference constant: the largest finite c of the evaluated components
+    int* comp_of;   // [rows] component at a position, -1 for none
+    float* illb;    // [Kpad] by component: > 0 for an ill-conditioned one
+    float* scra;    // [Kpad] by component: bound of the error of its approximate log2 z at the centre ...
+    float* scrw;    // [Kpad] ... and per unit of |x - g|^2
+    int* flags;     // [8]: [0] any ill-conditioned component, [4] how many, [2] slots of the list, [5] slots of its first
+                    //      kind, [6] evaluated components (positions [0, flags[6])); [1], [3], [7]: see launch_cand_count_wide
     int* ill_list;  // [WIDE_MAX_ILL] ascending indices of the ill-conditioned components
     float* mu_c;    // [WIDE_MAX_ILL][D] their means, packed: the sub-mixture the FP32 kernels evaluate exactly
     float* w2_c;    // [WIDE_MAX_ILL][D] their weights (log2 e / 2) / var
@@ -48,19 +57,27 @@ struct WideBuffers {
     float* top;     // [WIDE_PIECE][4] per point: its two largest approximate log2 z - c_ref and their components
     float* partial; // [R * CL][pcols][128] per-CTA partial statistics of the second sweep
     double* llpart; // [WIDE_LL_BLOCKS] partial sums of log Z
+    // Screening of the (point, ill-conditioned component) pairs by sweep 1 and their exact evaluation pair by pair:
+    float* scr;     // [rows] pairs: (c - c_ref + error allowance, allowance per unit of |x - g|^2); -inf for the others
+    int* slot_of;   // [rows] slot in the list of the component at a position, -1 if it is not listed
+    int* scr_mask;  // [rows / 32] nonzero where a chunk of 32 positions holds a listed component
+    float* n2;      // [WIDE_PIECE] |x_i - g|^2
+    unsigned* cand; // [WIDE_PIECE][words] bit (i, slot): the pair may matter (set by sweep 1)
+    unsigned* candT;// [WIDE_MAX_ILL][WIDE_CANDT_WORDS] bit (slot, i): the pair matters (set by the exact evaluation)
+    int* ctl;       // [8]: [0] pairs sweep 1 let through, [1] nonzero: too many, the FP32 kernels evaluate the sub-mixture
+                    //      densely, [2] nonzero: the pairs are evaluated one by one, [3] pairs that mattered
 };
 
 bool wide_supports(int D, int K);
 WidePlan wide_plan(int D, int K, int num_sms);
-// flags are cleared, then: scales, coefficient planes, constants; components whose error estimate exceeds cond_limit or
-// whose weight pi_k is below min_weight are flagged (flags[4] counts them) and excluded from the tensor passes (c = -inf).
+// flags are cleared, then: scales; components whose error estimate exceeds cond_limit or whose weight pi_k is below
+// min_weight are flagged (flags[4] counts them), listed (flags[2], flags[5]) and placed behind the others (flags[6] =
+// how many the tensor passes evaluate); coefficient planes and constants by position.
 cudaError_t launch_prepare_wide(cudaStream_t s, int D, int K, const float* pi, const float* mu, const float* var,
                                 const WideBuffers& wb, float cond_limit, float min_weight);
 // n <= WIDE_PIECE points: X -> the fp16 planes of Y (rows up to the next multiple of 256 are written as zeros).
 cudaError_t launch_transform_wide(cudaStream_t s, const float* X, int64_t n, int D, const WideBuffers& wb, int* status);
-// The components flagged by launch_prepare_wide: their list (flags[2] = how many), then their rows of the FP32 path's
-// derived parameters packed into wb.mu_c / w2_c / c2d_c.
-cudaError_t launch_ill_list_wide(cudaStream_t s, int D, int K, const WideBuffers& wb);
+// The listed components' rows of the FP32 path's derived parameters packed into wb.mu_c / w2_c / c2d_c.
 cudaError_t launch_ill_gather_wide(cudaStream_t s, int D, int n_ill, const WideBuffers& wb, const float* mu, const float* w2,
                                    const double* c2d);
 // wb.logz_x = wb.logz corrected by the exact values of every point's two leading terms (mu, w2, c2d: the FP32 path's
@@ -73,12 +90,33 @@ cudaError_t launch_merge_ll_wide(cudaStream_t s, int64_t n, const WideBuffers& w
 // stats rows of the listed components += wb.stats_c.
 cudaError_t launch_ill_scatter_wide(cudaStream_t s, int D, int K, int n_ill, const WideBuffers& wb, double* Nk, double* S1,
                                     double* S2);
-// First sweep over the n points whose planes were written: log2 Z per point (over the well-conditioned components) -> wb.logz.
-cudaError_t launch_lse_wide(cudaStream_t s, int64_t n, int D, int K, const WideBuffers& wb, int num_sms, int* status);
+// wb.flags[1] += wb.ctl[0] (pairs marked), wb.flags[3] += wb.ctl[3] (pairs kept), wb.flags[7] += 1 if the piece went through
+// the dense kernels: totals of a step, for diagnostics.
+cudaError_t launch_cand_count_wide(cudaStream_t s, const WideBuffers& wb);
+// First sweep over the n points whose planes were written: log2 Z per point over the Kg evaluated components -> wb.logz.
+// n_listed > 0 (listed components, n_slots slots of the list): the sweep also marks in wb.cand every pair of a point and a
+// listed component whose approximate log2 z, raised by its error bound, comes within 2^-40 of the point's maximum, and
+// counts the marks in wb.ctl[0]; wb.n2, wb.cand (zeroed) and wb.ctl (zeroed) must have been prepared for the piece.
+cudaError_t launch_lse_wide(cudaStream_t s, int64_t n, int D, int K, int Kg, int n_listed, int n_slots, const WideBuffers& wb,
+                            int num_sms, int* status);
+// wb.n2[i] = |x_i - g|^2 for the n points of a piece.
+cudaError_t launch_norm_wide(cudaStream_t s, const float* X, int64_t n, int D, const WideBuffers& wb);
+// Clears wb.ctl, the n rows of wb.cand and the n_slots rows of wb.candT before a piece's first sweep.
+cudaError_t launch_cand_clear_wide(cudaStream_t s, int64_t n, int n_slots, const WideBuffers& wb);
+// After sweep 1: wb.ctl[1] = (wb.ctl[0] > max_pairs), wb.ctl[2] = !wb.ctl[1].
+cudaError_t launch_cand_gate_wide(cudaStream_t s, const WideBuffers& wb, long long max_pairs);
+// The marked pairs evaluated exactly, one warp per point (no-op when wb.ctl[1] is set): logz_ill[i] = log2 of the sum of
+// the listed components' exact densities at point i over the pairs that reach 2^-40 of wb.logz[i] (-inf if none); those
+// pairs are marked in wb.candT.
+cudaError_t launch_cand_lse_wide(cudaStream_t s, const float* X, int64_t n, int D, int n_slots, const WideBuffers& wb,
+                                 double* logz_ill);
+// wb.stats_c += the statistics of the pairs marked in wb.candT with r = 2^(exact log2 z - wb.logz_x[i]); one block per
+// slot, points in ascending order (no-op when wb.ctl[1] is set).
+cudaError_t launch_cand_mstep_wide(cudaStream_t s, const float* X, int64_t n, int D, int n_slots, const WideBuffers& wb);
 // Second sweep: responsibilities from wb.logz, statistics accumulated into wb.partial (+=).
-cudaError_t launch_em_wide(cudaStream_t s, int64_t n, int D, int K, const WideBuffers& wb, int num_sms, int* status);
+cudaError_t launch_em_wide(cudaStream_t s, int64_t n, int D, int K, int Kg, const WideBuffers& wb, int num_sms, int* status);
 // stats += the partial blocks (fixed order, float64, scale / centre / column order undone).
-cudaError_t launch_reduce_wide(cudaStream_t s, int D, int K, const WideBuffers& wb, int num_sms, double* Nk, double* S1,
-                               double* S2);
+cudaError_t launch_reduce_wide(cudaStream_t s, int D, int K, int Kg, const WideBuffers& wb, int num_sms, double* Nk,
+                               double* S1, double* S2);
 
 }  // namespace fg

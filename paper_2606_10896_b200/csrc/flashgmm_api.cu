@@ -34,7 +34,7 @@ struct ScratchLayout {
     size_t tc_phi, tc_plo, tc_tk, tc_ck, tc_sd, tc_kap, tc_gd, tc_illb, tc_flags, tc_xg, tc_xl, tc_partial, tc_llpart, tc_partial_bytes, tc_yhi, tc_ylo, tc_phirm, tc_plorm, tc_tkck, tc_illlist, tc_illcache, tc_decdim, tc_decw, tc_decmu;
     bool tc;
     // the tensor-core path for D > 128
-    size_t w_sd, w_kap, w_gd, w_phi, w_plo, w_tk, w_tkck, w_ckd, w_cref, w_illb, w_flags, w_yhi, w_ylo, w_logz, w_partial, w_llpart, w_illlist, w_muc, w_w2c, w_c2dc, w_statsc, w_top, w_logzx;
+    size_t w_sd, w_kap, w_gd, w_phi, w_plo, w_tk, w_tkck, w_ckd, w_cref, w_illb, w_flags, w_yhi, w_ylo, w_logz, w_partial, w_llpart, w_illlist, w_muc, w_w2c, w_c2dc, w_statsc, w_top, w_logzx, w_compof, w_scra, w_scrw, w_scr, w_slotof, w_scrmask, w_n2, w_cand, w_candT, w_ctl;
     size_t w_partial_bytes;
     bool wide;
 };
@@ -89,6 +89,7 @@ ScratchLayout scratch_layout(int D, int K, bool planes) {
         L.tc_ylo = take(TC_YPLANE_BYTES);
     }
     L.w_sd = L.w_kap = L.w_gd = L.w_phi = L.w_plo = L.w_tk = L.w_tkck = L.w_ckd = L.w_cref = L.w_illb = L.w_flags = L.w_yhi = L.w_ylo = L.w_logz = L.w_partial = L.w_llpart = L.w_illlist = L.w_muc = L.w_w2c = L.w_c2dc = L.w_statsc = L.w_top = L.w_logzx = 0;
+    L.w_compof = L.w_scra = L.w_scrw = L.w_scr = L.w_slotof = L.w_scrmask = L.w_n2 = L.w_cand = L.w_candT = L.w_ctl = 0;
     L.w_partial_bytes = 0;
     L.wide = wide_supports(D, K) && planes;
     if (L.wide) {
@@ -96,14 +97,24 @@ ScratchLayout scratch_layout(int D, int K, bool planes) {
         L.w_sd = take((size_t)wp.Dpad * 4);
         L.w_kap = take((size_t)wp.Dpad * 4);
         L.w_gd = take((size_t)wp.Dpad * 4);
-        L.w_phi = take((size_t)wp.Kpad * wp.Dpad * 4);
-        L.w_plo = take((size_t)wp.Kpad * wp.Dpad * 4);
-        L.w_tk = take((size_t)wp.Kpad * 4);
-        L.w_tkck = take((size_t)wp.Kpad * 8);
-        L.w_ckd = take((size_t)wp.Kpad * 8);
+        L.w_phi = take((size_t)wp.rows * wp.Dpad * 4);
+        L.w_plo = take((size_t)wp.rows * wp.Dpad * 4);
+        L.w_tk = take((size_t)wp.rows * 4);
+        L.w_tkck = take((size_t)wp.rows * 8);
+        L.w_ckd = take((size_t)wp.rows * 8);
         L.w_cref = take(8);
         L.w_illb = take((size_t)wp.Kpad * 4);
         L.w_flags = take(32);
+        L.w_compof = take((size_t)wp.rows * 4);
+        L.w_scra = take((size_t)wp.Kpad * 4);
+        L.w_scrw = take((size_t)wp.Kpad * 4);
+        L.w_scr = take((size_t)wp.rows * 8);
+        L.w_slotof = take((size_t)wp.rows * 4);
+        L.w_scrmask = take((size_t)wp.rows / 32 * 4);
+        L.w_n2 = take((size_t)WIDE_PIECE * 4);
+        L.w_cand = take((size_t)WIDE_PIECE * WIDE_CAND_WORDS * 4);
+        L.w_candT = take((size_t)WIDE_MAX_ILL * WIDE_CANDT_WORDS * 4);
+        L.w_ctl = take(32);
         L.w_logz = take((size_t)WIDE_PIECE * 8);
         L.w_top = take((size_t)WIDE_PIECE * 16);
         L.w_logzx = take((size_t)WIDE_PIECE * 8);
@@ -158,6 +169,9 @@ struct gmm_ctx {
     int wide_n_first = 0;            // of which the first kind (flagged by the error estimate: mostly collapsed components)
     int wide_n_list = 0;             // slots of the packed sub-mixture (the ill-conditioned components plus padding)
     int wide_n_ill = 0;              // ill-conditioned components of the current step on the D > 128 tensor path
+    int wide_n_good = 0;             // components the tensor passes evaluate in the current step (the others are listed)
+    int wide_sparse = 1;             // GMM_WIDE_SPARSE: 0 = the listed components always go through the dense FP32 kernels,
+                                     // 1 = pair by pair unless sweep 1 marks too many pairs, 2 = always pair by pair (tests)
     int tc_n_ill = 0;                // ill-conditioned components at the last result that was read back (picks the filter)
     int tc_force_filter = -1;        // GMM_TC_FILTER=plain / tight: 0 / 1 (tests); -1: automatic
     int sticky_status = 0;           // status bits read off the device but not yet reported (see ensure_scratch)
@@ -238,6 +252,16 @@ struct gmm_ctx {
         b.w2_c = reinterpret_cast<float*>(scratch + lay.w_w2c);
         b.c2d_c = reinterpret_cast<double*>(scratch + lay.w_c2dc);
         b.stats_c = reinterpret_cast<double*>(scratch + lay.w_statsc);
+        b.comp_of = reinterpret_cast<int*>(scratch + lay.w_compof);
+        b.scra = reinterpret_cast<float*>(scratch + lay.w_scra);
+        b.scrw = reinterpret_cast<float*>(scratch + lay.w_scrw);
+        b.scr = reinterpret_cast<float*>(scratch + lay.w_scr);
+        b.slot_of = reinterpret_cast<int*>(scratch + lay.w_slotof);
+        b.scr_mask = reinterpret_cast<int*>(scratch + lay.w_scrmask);
+        b.n2 = reinterpret_cast<float*>(scratch + lay.w_n2);
+        b.cand = reinterpret_cast<unsigned*>(scratch + lay.w_cand);
+        b.candT = reinterpret_cast<unsigned*>(scratch + lay.w_candT);
+        b.ctl = reinterpret_cast<int*>(scratch + lay.w_ctl);
         return b;
     }
 };
@@ -391,21 +415,21 @@ int prepare_and_choose(gmm_ctx* ctx, int64_t N, int D, int K, const float* pi, c
         if (limit < 0.f) limit = ctx->tc_cond_scale * std::sqrt((float)((double)N / (double)K));
         const WideBuffers wb = ctx->wide();
         KL(launch_prepare_wide(ctx->stream, D, K, pi, mu, var, wb, limit, (float)((double)ctx->wide_min_points / (double)N)));
-        ctx->launches += 2;
-        int n_ill = 0;
-        CU(cudaMemcpyAsync(&n_ill, wb.flags + 4, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
+        ctx->launches += 4;
+        // how many components were flagged, the length of their list and how many are left to the tensor passes: one
+        // small synchronisation per step, against seconds of compute at these shapes
+        int fl[8];
+        CU(cudaMemcpyAsync(fl, wb.flags, sizeof(fl), cudaMemcpyDeviceToHost, ctx->stream));
         CU(cudaStreamSynchronize(ctx->stream));
+        const int n_ill = fl[4];
         ctx->wide_n_ill = n_ill;
+        ctx->wide_n_good = fl[6];
         if (n_ill + 64 > WIDE_MAX_ILL || 2 * n_ill > K) return GMM_OK;     // too many: the FP32 kernels take the whole step
         if (n_ill > 0) {
-            // The flagged components take no part in the tensor passes; the FP32 kernels evaluate them exactly as a packed
-            // sub-mixture (a collapsed component is hopeless for every point but its own, which those kernels notice after
-            // the first 32 dimensions of a tile).
-            KL(launch_ill_list_wide(ctx->stream, D, K, wb));
-            // (the list has a gap of empty slots between its two kinds of components: its length comes back with it)
-            int fl[8];
-            CU(cudaMemcpyAsync(fl, wb.flags, sizeof(fl), cudaMemcpyDeviceToHost, ctx->stream));
-            CU(cudaStreamSynchronize(ctx->stream));
+            // The flagged components take no part in the tensor passes: they are evaluated exactly as a packed sub-mixture,
+            // pair by pair where sweep 1 finds that a pair can matter, or densely by the FP32 kernels (a collapsed component
+            // is hopeless for every point but its own, which those kernels notice after the first 32 dimensions of a tile).
+            // (the list has a gap of empty slots between its two kinds of components)
             const int n_list = fl[2];
             ctx->wide_n_list = n_list;
             ctx->wide_n_first = fl[5] < n_list ? fl[5] : n_list;
@@ -464,34 +488,51 @@ int accumulate_points(gmm_ctx* ctx, int path, const float* X, int64_t n, int D, 
             CU(cudaMemsetAsync(wb.stats_c, 0, ((size_t)n_ill + 2 * (size_t)n_ill * D) * sizeof(double), ctx->stream));
         }
         CU(cudaMemsetAsync(wb.llpart, 0, 256 * 8, ctx->stream));
+        const int Kg = ctx->wide_n_good;
+        const int n_listed = n_ill > 0 ? ctx->wide_n_ill : 0;
+        const bool screen = n_ill > 0 && ctx->wide_sparse != 0;
+        const int* dense_if = screen ? wb.ctl + 1 : nullptr;             // the dense kernels run when the gate says so
         for (int64_t off = 0; off < n; off += ctx->wide_piece) {
             const int64_t cnt = (n - off < ctx->wide_piece) ? (n - off) : ctx->wide_piece;
             const float* Xs = X + off * D;
             CU(cudaMemsetAsync(wb.partial, 0, ctx->lay.w_partial_bytes, ctx->stream));
+            if (screen) {
+                CU(launch_cand_clear_wide(ctx->stream, cnt, n_ill, wb));
+                KL(launch_norm_wide(ctx->stream, Xs, cnt, D, wb));
+            }
             CHECK(prof_begin(ctx));
             KL(launch_transform_wide(ctx->stream, Xs, cnt, D, wb, &ctx->result()->status));
-            KL(launch_lse_wide(ctx->stream, cnt, D, K, wb, ctx->sms, &ctx->result()->status));
+            KL(launch_lse_wide(ctx->stream, cnt, D, K, Kg, screen ? n_listed : 0, n_ill, wb, ctx->sms, &ctx->result()->status));
             if (ctx->wide_refine) KL(launch_refine_wide(ctx->stream, Xs, cnt, D, K, mu, ctx->w2(), ctx->c2d(), wb));
             else CU(cudaMemcpyAsync(wb.logz_x, wb.logz, (size_t)cnt * 8, cudaMemcpyDeviceToDevice, ctx->stream));
-            if (n_ill > 0)
-                KL(launch_lse_fp32(ctx->stream, Xs, cnt, D, n_ill, wb.mu_c, wb.w2_c, wb.c2d_c, ctx->center(), ctx->logZ2(), nullptr, wb.logz));
+            if (n_ill > 0) {
+                if (screen) {
+                    // more than one pair in 64 marked (or the pair-by-pair route switched off): the dense kernels are cheaper
+                    const long long max_pairs = ctx->wide_sparse >= 2 ? ((long long)1 << 62) : (long long)cnt * n_ill / 64;
+                    KL(launch_cand_gate_wide(ctx->stream, wb, max_pairs));
+                    KL(launch_cand_lse_wide(ctx->stream, Xs, cnt, D, n_ill, wb, ctx->logZ2()));
+                }
+                KL(launch_lse_fp32(ctx->stream, Xs, cnt, D, n_ill, wb.mu_c, wb.w2_c, wb.c2d_c, ctx->center(), ctx->logZ2(), nullptr, wb.logz, dense_if));
+            }
             KL(launch_merge_ll_wide(ctx->stream, cnt, wb, n_ill > 0 ? ctx->logZ2() : nullptr));
-            KL(launch_em_wide(ctx->stream, cnt, D, K, wb, ctx->sms, &ctx->result()->status));
+            KL(launch_em_wide(ctx->stream, cnt, D, K, Kg, wb, ctx->sms, &ctx->result()->status));
             CHECK(prof_end(ctx));
-            KL(launch_reduce_wide(ctx->stream, D, K, wb, ctx->sms, Nk, S1, S2));
+            KL(launch_reduce_wide(ctx->stream, D, K, Kg, wb, ctx->sms, Nk, S1, S2));
             if (n_ill > 0) {
                 double* Nk_c = wb.stats_c;
                 double* S1_c = Nk_c + n_ill;
                 double* S2_c = S1_c + (size_t)n_ill * D;
+                if (screen) KL(launch_cand_mstep_wide(ctx->stream, Xs, cnt, D, n_ill, wb));
                 if (n_a > 0) {
-                    KL(launch_mstep_fp32(ctx->stream, Xs, cnt, D, n_a, wb.mu_c, wb.w2_c, wb.c2d_c, ctx->center(), wb.logz_x, ctx->partials(), plan_a, true));
+                    KL(launch_mstep_fp32(ctx->stream, Xs, cnt, D, n_a, wb.mu_c, wb.w2_c, wb.c2d_c, ctx->center(), wb.logz_x, ctx->partials(), plan_a, true, dense_if));
                     KL(launch_reduce_partials(ctx->stream, D, n_a, plan_a.splits, ctx->partials(), ctx->center(), Nk_c, S1_c, S2_c, true));
                 }
                 if (n_b > 0) {
                     const size_t o = (size_t)n_a * D;
-                    KL(launch_mstep_fp32(ctx->stream, Xs, cnt, D, n_b, wb.mu_c + o, wb.w2_c + o, wb.c2d_c + n_a, ctx->center(), wb.logz_x, ctx->partials(), plan_b, true));
+                    KL(launch_mstep_fp32(ctx->stream, Xs, cnt, D, n_b, wb.mu_c + o, wb.w2_c + o, wb.c2d_c + n_a, ctx->center(), wb.logz_x, ctx->partials(), plan_b, true, dense_if));
                     KL(launch_reduce_partials(ctx->stream, D, n_b, plan_b.splits, ctx->partials(), ctx->center(), Nk_c + n_a, S1_c + o, S2_c + o, true));
                 }
+                if (screen) KL(launch_cand_count_wide(ctx->stream, wb));
             }
         }
         if (n_ill > 0) KL(launch_ill_scatter_wide(ctx->stream, D, K, n_ill, wb, Nk, S1, S2));
@@ -608,6 +649,7 @@ int gmm_create(gmm_ctx** out, int device, void* cuda_stream) {
     if (const char* e = std::getenv("GMM_TC_FLUSH")) ctx->tc_flush = std::atoi(e);
     if (const char* e = std::getenv("GMM_WIDE_MIN_POINTS")) ctx->wide_min_points = std::atof(e);
     if (const char* e = std::getenv("GMM_WIDE_REFINE")) ctx->wide_refine = std::atoi(e) != 0;
+    if (const char* e = std::getenv("GMM_WIDE_SPARSE")) ctx->wide_sparse = std::atoi(e);
     if (const char* e = std::getenv("GMM_WIDE_PIECE")) {
         const long long v = std::atoll(e);
         if (v >= 256 && v <= WIDE_PIECE) ctx->wide_piece = v / 256 * 256;
@@ -670,6 +712,20 @@ int gmm_last_exact_count(const gmm_ctx* ctx) {
     if (!ctx) return GMM_EINVAL;
     if (ctx->last_path != GMM_PATH_TENSOR) return 0;
     return wide_supports(ctx->capD, ctx->capK) ? ctx->wide_n_ill : ctx->tc_n_ill;
+}
+
+int gmm_last_exact_pairs(gmm_ctx* ctx, int64_t* marked, int64_t* kept, int* dense_pieces) {
+    if (!ctx || !marked || !kept || !dense_pieces) return GMM_EINVAL;
+    *marked = *kept = 0;
+    *dense_pieces = 0;
+    if (ctx->last_path != GMM_PATH_TENSOR || !wide_supports(ctx->capD, ctx->capK) || !ctx->lay.wide || ctx->wide_n_ill <= 0) return GMM_OK;
+    int fl[8];
+    CU(cudaMemcpyAsync(fl, ctx->wide().flags, sizeof(fl), cudaMemcpyDeviceToHost, ctx->stream));
+    CU(cudaStreamSynchronize(ctx->stream));
+    *marked = fl[1];
+    *kept = fl[3];
+    *dense_pieces = fl[7];
+    return GMM_OK;
 }
 
 int gmm_em_step(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const float* pi, const float* mu,

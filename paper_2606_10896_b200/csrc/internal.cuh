@@ -39,13 +39,15 @@ cudaError_t launch_center_fp32(cudaStream_t s, int D, int K, const float* mu, fl
 // tiles whose terms all lie 2^-40 below it are not evaluated to the end (their terms count as zero).
 cudaError_t launch_lse_fp32(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu,
                             const float* w2, const double* c2d, const float* g, double* logZ2, double* llpart,
-                            const double* lower2 = nullptr);
+                            const double* lower2 = nullptr, const int* run_if = nullptr);
 // out[i] = ln 2 * logZ2[i]: the per-point log-density in natural units, fp32
 cudaError_t launch_logz_out_fp32(cudaStream_t s, const double* logZ2, int64_t n, float* out);
 cudaError_t launch_mstep_fp32(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu,
                               const float* w2, const double* c2d, const float* g, const double* logZ2, float* partials,
-                              const Fp32Plan& plan, bool early = false);
+                              const Fp32Plan& plan, bool early = false, const int* run_if = nullptr);
 // early (D > 128 only): skip the tiles in which no responsibility can reach 2^-40 (sub-mixtures of collapsed components)
+// run_if (launch_lse_fp32, and launch_mstep_fp32 for D > 128): NULL, or a device flag: the kernel does nothing unless
+// run_if[0] != 0 (the partials of a gated-off M-step stay zero).
 // run_if: NULL, or a device flag: the kernel does nothing unless run_if[0] != 0.
 // gather: NULL, or device row indices: the points are X[gather[0 .. min(n, *gather_count))], and the outputs go to those
 // rows of idx / resp (n then bounds the number of gathered points, and sizes the grid).

@@ -28,6 +28,8 @@ EXPORTS = {
     "gmm_set_path": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int]),
     "gmm_last_path": (ctypes.c_int, [ctypes.c_void_p]),
     "gmm_last_exact_count": (ctypes.c_int, [ctypes.c_void_p]),
+    "gmm_last_exact_pairs": (ctypes.c_int, [ctypes.c_void_p, ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int64),
+                                            ctypes.POINTER(ctypes.c_int)]),
     "gmm_tensor_path_supports": (ctypes.c_int, [ctypes.c_int, ctypes.c_int]),
     "gmm_auto_path": (ctypes.c_int, [ctypes.c_int, ctypes.c_int]),
     "gmm_em_step": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_int,
@@ -206,6 +208,12 @@ class Context:
 
     def gmm_last_exact_count(self) -> int:
         return int(lib.gmm_last_exact_count(self._h))
+
+    def gmm_last_exact_pairs(self):
+        """(marked, kept, dense_pieces) of the most recent wide tensor-path step: see include/flashgmm.h."""
+        a, b, c = ctypes.c_int64(0), ctypes.c_int64(0), ctypes.c_int(0)
+        self._check(lib.gmm_last_exact_pairs(self._h, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c)))
+        return int(a.value), int(b.value), int(c.value)
 
     def gmm_launch_count(self) -> int:
         return int(lib.gmm_launch_count(self._h))

@@ -170,3 +170,48 @@ def test_wide_data_far_from_the_origin(fg, ctx):
     mu = (mu + 200.0).astype(np.float32)
     ctx.gmm_set_path(fg.GMM_PATH_TENSOR)
     _step_and_check(fg, ctx, X, pi, mu, var, "wide, 200 units from the origin")
+
+
+def _with_listed_components(rng, N, D, K, sep=0.3):
+    X, pi, mu, var = _clustered(rng, N, D, K, sep=sep)
+    for j in range(5):                       # collapsed onto a point
+        mu[j] = X[50 + j]
+        var[j] = 1e-6
+    pi[8:14] = 2e-4                          # light, broad
+    pi = (pi / pi.sum()).astype(np.float32)
+    return X, pi, mu, var
+
+
+@pytest.mark.parametrize("mode", ["0", "1", "2"])
+def test_listed_components_pair_by_pair_or_densely(fg, monkeypatch, mode):
+    """The components the tensor passes leave out are evaluated exactly either pair by pair (the pairs the first sweep
+    could not rule out: GMM_WIDE_SPARSE=2 always, 1 = the default when they are few) or by the FP32 kernels over the whole
+    sub-mixture (0); all three match the oracle, and the counters say which route ran."""
+    monkeypatch.setenv("GMM_WIDE_SPARSE", mode)
+    monkeypatch.setenv("GMM_WIDE_PIECE", "8192")
+    X, pi, mu, var = _with_listed_components(np.random.default_rng(31), 20_000, 288, 80)
+    with fg.Context(0) as c:
+        c.gmm_set_path(fg.GMM_PATH_TENSOR)
+        a = _step_and_check(fg, c, X, pi, mu, var, f"listed components, GMM_WIDE_SPARSE={mode}")
+        assert c.gmm_last_path() == fg.GMM_PATH_TENSOR and c.gmm_last_exact_count() >= 11
+        marked, kept, dense = c.gmm_last_exact_pairs()
+        if mode == "0":
+            assert (marked, kept, dense) == (0, 0, 0)
+        else:
+            # every collapsed component keeps its own point, a light one its cluster (about 250 points)
+            assert dense == 0 and kept >= 5 + 6 * 100 and marked >= kept and marked < 20 * kept
+        Nk, S1, S2, _ = c.gmm_em_step(_t(X), _t(pi), _t(mu), _t(var))
+        for u, v in zip(a, (Nk, S1, S2)):
+            assert np.array_equal(u, v.cpu().numpy())            # same bits in a second run
+
+
+def test_many_marked_pairs_go_to_the_dense_kernels(fg, ctx):
+    """Clusters that overlap almost completely: every point is a candidate for every light component, more than one pair
+    in 64 is marked, and the step hands the sub-mixture of those pieces to the FP32 kernels."""
+    X, pi, mu, var = _clustered(np.random.default_rng(37), 24_000, 256, 64, sep=0.01)
+    pi[3:9] = 5e-4
+    pi = (pi / pi.sum()).astype(np.float32)
+    ctx.gmm_set_path(fg.GMM_PATH_TENSOR)
+    _step_and_check(fg, ctx, X, pi, mu, var, "overlapping clusters, light components")
+    marked, kept, dense = ctx.gmm_last_exact_pairs()
+    assert ctx.gmm_last_exact_count() >= 6 and dense == 1 and marked > 24_000 * 6 // 64

@@ -60,10 +60,12 @@ struct LseParams {
     const double* cref;
     double* logz;
     double* llpart;
-    float4* top;         // [n] per point: its two largest approximate log2 z (relative to c_ref) and their components
+    float* top;          // [n][2 NTOP] per point: its NTOP largest approximate log2 z (relative to c_ref), then their positions
     int* status;
     // screening of the listed (ill-conditioned) components, all NULL / 0 when there are none
-    const float2* scr;   // [NC * 128] (c_k - c_ref + allowance, allowance per unit of |x - g|^2); -inf for unlisted components
+    bool screen;         // listed components follow the evaluated ones and are screened
+    const float2* scr;   // [NC * 128] listed components: (c - c_ref + error allowance, allowance per unit of |x - g|^2);
+                         // evaluated components: (error allowance, allowance per unit of |x - g|^2)
     const int* scr_mask; // [NC * 4] nonzero where a chunk of 32 components holds a listed one
     const int* slot_of;  // [NC * 128]
     const float* n2;     // [n]
@@ -73,6 +75,30 @@ struct LseParams {
     int* ctl;
 };
 
+// NTOP: how many of a point's largest approximate log2 z the sweep reports (2 for the EM step's exact normaliser, m + 2 for
+// the top-m assignment).
+template <int NTOP>
+struct WideTop {
+    float a[NTOP];
+    int i[NTOP];
+    __device__ __forceinline__ void init() {
+#pragma unroll
+        for (int j = 0; j < NTOP; ++j) { a[j] = -CUDART_INF_F; i[j] = -1; }
+    }
+    __device__ __forceinline__ void insert(float val, int id) {      // descending; a later equal value stays behind
+        if (!(val > a[NTOP - 1])) return;
+        a[NTOP - 1] = val; i[NTOP - 1] = id;
+#pragma unroll
+        for (int j = NTOP - 1; j > 0; --j) {
+            if (a[j] > a[j - 1]) {
+                const float fv = a[j]; a[j] = a[j - 1]; a[j - 1] = fv;
+                const int fi = i[j]; i[j] = i[j - 1]; i[j - 1] = fi;
+            }
+        }
+    }
+};
+
+template <int NTOP>
 __global__ void __launch_bounds__(WT_THREADS, 1)
 lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, const __grid_constant__ CUtensorMap tm_ylo,
                 const __grid_constant__ CUtensorMap tm_phi, const __grid_constant__ CUtensorMap tm_plo) {
@@ -84,7 +110,7 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
     volatile int* drain_flag = &drain_s;
     float2* merge_s = reinterpret_cast<float2*>(smem + L_MERGE);
     double* ll_s = reinterpret_cast<double*>(smem + L_MERGE);      // after the last tile
-    __shared__ float4 top_s[128];
+    __shared__ float top_s[128][2 * NTOP + 1];
     __shared__ float xm_s[256];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -126,14 +152,14 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
         for (int64_t i = 0; i < ntl; ++i) {
             const int64_t row = (blockIdx.x + i * gridDim.x) * WIDE_TILE + pt;
             float m_run = -1e30f, s_run = 0.f;               // finite start: blocks of -inf logits must not make NaN
-            const float nrm = (p.scr != nullptr && row < p.n) ? __ldg(p.n2 + row) : 0.f;
+            const float nrm = ((p.screen || NTOP > 2) && row < p.n) ? __ldg(p.n2 + row) : 0.f;
             float thr_base = -1e30f;
             int nhit = 0;
-            float t1 = -CUDART_INF_F, t2 = -CUDART_INF_F;    // the two largest logits of this thread's chunks, and where
-            int i1 = -1, i2 = -1;
+            WideTop<NTOP> tl;                                // the largest logits of this thread's chunks, and where
+            tl.init();
             for (int g = 0; g < NG; ++g) {
                 const int nch = (NC - 2 * g < 2) ? (NC - 2 * g) : 2;
-                const bool screening = p.scr != nullptr && g >= p.scr_group;
+                const bool screening = p.screen && g >= p.scr_group;
                 if (screening && g == p.scr_group) {          // the two warpgroups' running maxima, merged once per tile
                     xm_s[grp * 128 + pt] = m_run;
                     named_bar_sync(3, 256);
@@ -193,12 +219,27 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
                                 s_run *= fast_ex2(m_run - bmax);
                                 m_run = bmax;
                             }
-                            if (bmax > t2) {                 // (rare after the first chunks)
+                            if (NTOP == 2) {
+                                if (bmax > tl.a[NTOP - 1]) { // (rare after the first chunks)
 #pragma unroll
-                                for (int j = 0; j < 32; ++j) {
-                                    if (l[j] > t2) {
-                                        if (l[j] > t1) { t2 = t1; i2 = i1; t1 = l[j]; i1 = col0 + j; }
-                                        else { t2 = l[j]; i2 = col0 + j; }
+                                    for (int j = 0; j < 32; ++j) tl.insert(l[j], col0 + j);
+                                }
+                            } else {
+                                // the assignment ranks by an UPPER bound of the exact value (approximate value + what it can be
+                                // wrong by for this point): what is not reported then lies below the last reported bound
+                                const float4* sc4 = reinterpret_cast<const float4*>(p.scr + col0);
+                                float bub = -CUDART_INF_F;
+#pragma unroll
+                                for (int j = 0; j < 32; j += 2) {
+                                    const float4 sq = __ldg(sc4 + (j >> 1));
+                                    bub = fmaxf(bub, fmaxf(l[j] + fmaf(sq.y, nrm, sq.x), l[j + 1] + fmaf(sq.w, nrm, sq.z)));
+                                }
+                                if (bub > tl.a[NTOP - 1]) {
+#pragma unroll
+                                    for (int j = 0; j < 32; j += 2) {
+                                        const float4 sq = __ldg(sc4 + (j >> 1));
+                                        tl.insert(l[j] + fmaf(sq.y, nrm, sq.x), col0 + j);
+                                        tl.insert(l[j + 1] + fmaf(sq.w, nrm, sq.z), col0 + j + 1);
                                     }
                                 }
                             }
@@ -219,27 +260,22 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
             // merge the two warpgroups' pairs; warpgroup 0 writes log2 Z and the two leading candidates
             if (grp == 1) {
                 merge_s[pt] = make_float2(m_run, s_run);
-                top_s[pt] = make_float4(t1, t2, __int_as_float(i1), __int_as_float(i2));
+#pragma unroll
+                for (int j = 0; j < NTOP; ++j) { top_s[pt][j] = tl.a[j]; top_s[pt][NTOP + j] = __int_as_float(tl.i[j]); }
             }
             named_bar_sync(1, 256);
             if (grp == 0) {
                 const float2 o = merge_s[pt];
                 const float m = fmaxf(m_run, o.x);
                 const float s = s_run * fast_ex2(m_run - m) + o.y * fast_ex2(o.x - m);
-                const float4 ot = top_s[pt];
-                const float ov[2] = {ot.x, ot.y};
-                const int oi[2] = {__float_as_int(ot.z), __float_as_int(ot.w)};
 #pragma unroll
-                for (int j = 0; j < 2; ++j) {
-                    if (ov[j] > t2) {
-                        if (ov[j] > t1) { t2 = t1; i2 = i1; t1 = ov[j]; i1 = oi[j]; }
-                        else { t2 = ov[j]; i2 = oi[j]; }
-                    }
-                }
+                for (int j = 0; j < NTOP; ++j) tl.insert(top_s[pt][j], __float_as_int(top_s[pt][NTOP + j]));
                 if (row < p.n && !*abort_flag) {
                     const double lz = cref + (double)m + (double)log2f(s);
                     p.logz[row] = lz;
-                    p.top[row] = make_float4(t1, t2, __int_as_float(i1), __int_as_float(i2));
+                    float* tp = p.top + row * (2 * NTOP);
+#pragma unroll
+                    for (int j = 0; j < NTOP; ++j) { tp[j] = tl.a[j]; tp[NTOP + j] = __int_as_float(tl.i[j]); }
                     ll_acc += lz;
                 }
             }
@@ -1027,7 +1063,8 @@ __global__ void __launch_bounds__(256) wide_prepare_kernel(int D, int Dpad, cons
 }
 
 // c_ref = the largest finite c among the positions the tensor passes evaluate; tkck[pos] = (t, c - c_ref) in fp32 (-inf
-// where the position takes no part); scr[pos] = (c - c_ref + scra, scrw) for a listed component, (-inf, 0) elsewhere.
+// where the position takes no part); scr[pos] = (c - c_ref + scra, scrw) for a listed component, (scra, scrw) for an
+// evaluated one, (-inf, 0) elsewhere.
 __global__ void __launch_bounds__(1024) wide_cref_kernel(int rows, const int* __restrict__ flags, const float* __restrict__ tk,
                                                          const double* __restrict__ ckd, const int* __restrict__ comp_of,
                                                          const int* __restrict__ slot_of, const float* __restrict__ scra,
@@ -1051,7 +1088,8 @@ __global__ void __launch_bounds__(1024) wide_cref_kernel(int rows, const int* __
         tkck[k] = make_float2(tk[k], in ? (float)(ckd[k] - r) : -CUDART_INF_F);
         const int c = comp_of[k];
         const bool listed = slot_of[k] >= 0 && c >= 0 && isfinite(ckd[k]);
-        scr[k] = listed ? make_float2((float)fmin(ckd[k] - r + (double)scra[c], 3e38), scrw[c]) : make_float2(-CUDART_INF_F, 0.f);
+        scr[k] = listed ? make_float2((float)fmin(ckd[k] - r + (double)scra[c], 3e38), scrw[c])
+                        : (in && c >= 0) ? make_float2(scra[c], scrw[c]) : make_float2(-CUDART_INF_F, 0.f);
     }
 }
 
@@ -1388,6 +1426,147 @@ __global__ void __launch_bounds__(256) wide_cand_mstep_kernel(const float* __res
     }
 }
 
+// ---- top-m assignment on wide data (paper Sections 4.2-4.3) -----------------------------------------------------------
+// Sweep 1 reports a point's NTOP evaluated components of largest UPPER BOUND (approximate log2 z plus what it can be wrong
+// by for that point; what is not reported lies below the last reported bound), its approximate log2 Z, and marks the listed
+// components that can matter for it.  One warp per point then evaluates exactly (a) the marked listed pairs, (b) the
+// reported candidates, in the order of their bounds, for as long as a bound reaches 2^-21 of the best exact value so far,
+// orders the exact values by (value, component) and writes the first m with r = 2^(log2 z - log2 Z'), Z' = Z with the
+// evaluated terms replaced by their exact values; places left over are filled from the reported candidates that were not
+// evaluated (their responsibilities are below 5e-7).  A point is left to the FP32 kernels (its row joins unc_rows) when
+// the answer is not certain: every reported candidate had to be evaluated and the m-th exact value does not clear the last
+// reported bound; fewer than m candidates exist; or (unless only indices are wanted) the terms that stay approximate make
+// up more than 1e-3 of Z'.
+struct WideAssignArgs {
+    const float* X; int64_t n; int D, K;
+    const float* mu; const float* w2; const double* c2d;      // the FP32 path's derived parameters, by component
+    const int* comp_of; const float* top; const double* logz; const double* cref; const float* n2;
+    const float* scra; const float* scrw;                     // error allowances by component
+    const unsigned* cand; int cand_words; const int* list; const float* mu_c; const float* w2_c; const double* c2d_c;
+    const int* ctl;
+    int m; int32_t* idx; float* resp; int32_t* unc_rows; int* unc_count; bool index_only;
+};
+
+template <int NTOP>
+__global__ void __launch_bounds__(256) wide_assign_refine_kernel(const WideAssignArgs g) {
+    if (g.ctl != nullptr && g.ctl[1] != 0) return;            // the piece went to the dense kernels as a whole
+    const int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (row >= g.n) return;
+    const int D = g.D, m = g.m;
+    const float* tp = g.top + row * (2 * NTOP);
+    float ub[NTOP];
+    int ap[NTOP];
+    int nvalid = 0;
+#pragma unroll
+    for (int j = 0; j < NTOP; ++j) {
+        ub[j] = __ldg(tp + j);
+        ap[j] = __float_as_int(__ldg(tp + NTOP + j));
+        if (ap[j] >= 0) ++nvalid;
+    }
+    const double lz = g.logz[row], cr = *g.cref;
+    const float nrm = __ldg(g.n2 + row);
+    const float* xr = g.X + row * D;
+    // exact values, the largest kept in order (value descending, component ascending)
+    double tv[GMM_MAX_TOPM];
+    int tk[GMM_MAX_TOPM];
+#pragma unroll
+    for (int j = 0; j < GMM_MAX_TOPM; ++j) { tv[j] = -CUDART_INF; tk[j] = -1; }
+    int n_exact = 0;
+    auto insert = [&](double val, int k) {
+        ++n_exact;
+        constexpr int L = GMM_MAX_TOPM - 1;
+        if (!(tk[L] < 0 || val > tv[L] || (val == tv[L] && k < tk[L]))) return;
+        tv[L] = val; tk[L] = k;
+#pragma unroll
+        for (int j = L; j > 0; --j) {
+            if (tk[j - 1] < 0 || tv[j] > tv[j - 1] || (tv[j] == tv[j - 1] && tk[j] < tk[j - 1])) {
+                const double fv = tv[j]; tv[j] = tv[j - 1]; tv[j - 1] = fv;
+                const int fi = tk[j]; tk[j] = tk[j - 1]; tk[j - 1] = fi;
+            }
+        }
+    };
+    // log2 Z' as a running (reference, sum): starts as Z itself; exact_part: the share of the exactly evaluated terms
+    double Mr = lz, Ss = (lz > -CUDART_INF) ? 1.0 : 0.0, exact_part = 0.0;
+    auto add_term = [&](double t) {
+        if (t > Mr) { const double f = exp2(Mr - t); Ss = Ss * f + 1.0; exact_part = exact_part * f + 1.0; Mr = t; }
+        else { const double e = exp2(t - Mr); Ss += e; exact_part += e; }
+    };
+    if (g.cand != nullptr) {
+        const double lim = lz - 40.0;
+        const int words = g.cand_words;
+        const unsigned b0 = (lane < words) ? g.cand[row * words + lane] : 0u;
+        const unsigned b1 = (lane + 32 < words) ? g.cand[row * words + 32 + lane] : 0u;
+        if (__any_sync(0xffffffffu, (b0 | b1) != 0u)) {
+            for (int wi = 0; wi < words; ++wi) {
+                unsigned word = __shfl_sync(0xffffffffu, wi < 32 ? b0 : b1, wi & 31);
+                while (word) {
+                    const int b = __ffs(word) - 1;
+                    word &= word - 1;
+                    const int slot = wi * 32 + b;
+                    const int k = __ldg(g.list + slot);
+                    if (k < 0) continue;
+                    const double l = wide_pair_log2z(xr, g.mu_c + (size_t)slot * D, g.w2_c + (size_t)slot * D, __ldg(g.c2d_c + slot), D, lane, lim);
+                    if (l >= lim && l > -CUDART_INF) { add_term(l); insert(l, k); }
+                }
+            }
+        }
+    }
+    int p = 0;                                                // reported candidates evaluated (a prefix)
+#pragma unroll
+    for (int j = 0; j < NTOP; ++j) {
+        // warp-uniform: the bounds descend, so the first that cannot matter ends the evaluation
+        if (j == p && ap[j] >= 0 && !(cr + (double)ub[j] < tv[0] - 21.0)) {
+            const int k = __ldg(g.comp_of + ap[j]);
+            if (k >= 0 && k < g.K) {
+                const double approx = cr + (double)(ub[j] - fmaf(__ldg(g.scrw + k), nrm, __ldg(g.scra + k)));
+                const double l = wide_pair_log2z(xr, g.mu + (size_t)k * D, g.w2 + (size_t)k * D, __ldg(g.c2d + k), D, lane, -CUDART_INF);
+                Ss -= exp2(approx - Mr);                      // its approximate term leaves the sum (Mr >= lz >= that term)
+                if (l > -CUDART_INF) { add_term(l); insert(l, k); }
+            }
+            ++p;
+        }
+    }
+    const int n_top = n_exact < GMM_MAX_TOPM ? n_exact : GMM_MAX_TOPM;
+    const int rest = nvalid - p;                              // reported candidates that were not evaluated (they do not matter)
+    bool certain = (n_top + rest >= m) && (Ss > 0.0) && (Ss < CUDART_INF);
+    if (certain && p == NTOP) {
+        // every reported candidate had to be evaluated: unreported components (all below the last bound) may matter too
+        double vm = tv[0];
+#pragma unroll
+        for (int j = 1; j < GMM_MAX_TOPM; ++j)
+            if (j == m - 1) vm = tv[j];
+        certain = n_top >= m && vm > cr + (double)ub[NTOP - 1];
+    }
+    if (certain && !g.index_only && !(Ss - exact_part <= 1e-3 * Ss)) certain = false;
+    if (!certain) {
+        if (lane == 0) g.unc_rows[atomicAdd(g.unc_count, 1)] = (int32_t)row;
+        return;
+    }
+    const double lzp = Mr + log2(Ss);
+    if (lane < m) {
+        double v;
+        int k;
+        if (lane < n_top) {
+            v = tv[0]; k = tk[0];
+#pragma unroll
+            for (int j = 1; j < GMM_MAX_TOPM; ++j)
+                if (lane == j) { v = tv[j]; k = tk[j]; }
+        } else {
+            const int q = p + (lane - n_top);                 // unevaluated candidates in the order of their bounds
+            float a = ub[0];
+            int pos = ap[0];
+#pragma unroll
+            for (int j = 1; j < NTOP; ++j)
+                if (q == j) { a = ub[j]; pos = ap[j]; }
+            k = __ldg(g.comp_of + pos);
+            v = cr + (double)(a - fmaf(__ldg(g.scrw + k), nrm, __ldg(g.scra + k)));
+        }
+        g.idx[row * m + lane] = k;
+        if (g.resp) g.resp[row * m + lane] = (float)exp2(v - lzp);
+    }
+}
+
 // The sub-mixture's statistics go to the rows of its components (which the tensor passes left at zero).
 __global__ void wide_ill_scatter_kernel(int D, int K, int n_ill, const int* __restrict__ list, const double* __restrict__ Nk_c,
                                         const double* __restrict__ S1_c, const double* __restrict__ S2_c, double* __restrict__ Nk,
@@ -1538,6 +1717,23 @@ cudaError_t launch_cand_mstep_wide(cudaStream_t s, const float* X, int64_t n, in
     return cudaGetLastError();
 }
 
+cudaError_t launch_assign_refine_wide(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu, const float* w2,
+                                      const double* c2d, int n_slots, bool screened, const WideBuffers& wb, int ntop, int m,
+                                      int32_t* idx, float* resp, int32_t* unc_rows, int* unc_count, bool index_only) {
+    if (m < 1 || m > GMM_MAX_TOPM || m > ntop) return cudaErrorInvalidValue;
+    WideAssignArgs g;
+    g.X = X; g.n = n; g.D = D; g.K = K; g.mu = mu; g.w2 = w2; g.c2d = c2d;
+    g.comp_of = wb.comp_of; g.top = wb.top; g.logz = wb.logz; g.cref = wb.cref; g.n2 = wb.n2; g.scra = wb.scra; g.scrw = wb.scrw;
+    g.cand = screened ? wb.cand : nullptr; g.cand_words = (n_slots + 31) / 32; g.list = wb.ill_list;
+    g.mu_c = wb.mu_c; g.w2_c = wb.w2_c; g.c2d_c = wb.c2d_c; g.ctl = screened ? wb.ctl : nullptr;
+    g.m = m; g.idx = idx; g.resp = resp; g.unc_rows = unc_rows; g.unc_count = unc_count; g.index_only = index_only;
+    const unsigned grid = (unsigned)((n + 7) / 8);
+    if (ntop == 6) wide_assign_refine_kernel<6><<<grid, 256, 0, s>>>(g);
+    else if (ntop == WIDE_MAX_TOP) wide_assign_refine_kernel<WIDE_MAX_TOP><<<grid, 256, 0, s>>>(g);
+    else return cudaErrorInvalidValue;
+    return cudaGetLastError();
+}
+
 cudaError_t launch_transform_wide(cudaStream_t s, const float* X, int64_t n, int D, const WideBuffers& wb, int* status) {
     if (n < 1 || n > WIDE_PIECE) return cudaErrorInvalidValue;
     const WidePlan pl = wide_plan(D, 1, 148);
@@ -1550,7 +1746,7 @@ cudaError_t launch_transform_wide(cudaStream_t s, const float* X, int64_t n, int
 }
 
 cudaError_t launch_lse_wide(cudaStream_t s, int64_t n, int D, int K, int Kg, int n_listed, int n_slots, const WideBuffers& wb,
-                            int num_sms, int* status) {
+                            int num_sms, int* status, int ntop) {
     if (n < 1 || n > WIDE_PIECE || Kg < 1 || Kg > K) return cudaErrorInvalidValue;
     const WidePlan pl = wide_plan(D, K, num_sms);
     const int64_t rp = rows_padded_of(n);
@@ -1561,7 +1757,11 @@ cudaError_t launch_lse_wide(cudaStream_t s, int64_t n, int D, int K, int Kg, int
     if (e == cudaSuccess) e = wide_make_map(&tm_ylo, wb.y_lo, rp, pitch, atoms, WIDE_TILE, 1);
     if (e == cudaSuccess) e = wide_make_map(&tm_phi, wb.p_hi, pl.rows, pitch, atoms, 128, 1);
     if (e == cudaSuccess) e = wide_make_map(&tm_plo, wb.p_lo, pl.rows, pitch, atoms, 128, 1);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(lse_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L_SMEM);
+    if (ntop != 2 && ntop != 6 && ntop != WIDE_MAX_TOP) return cudaErrorInvalidValue;
+    if (e == cudaSuccess)
+        e = ntop == 2 ? cudaFuncSetAttribute(lse_wide_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, L_SMEM)
+          : ntop == 6 ? cudaFuncSetAttribute(lse_wide_kernel<6>, cudaFuncAttributeMaxDynamicSharedMemorySize, L_SMEM)
+                      : cudaFuncSetAttribute(lse_wide_kernel<WIDE_MAX_TOP>, cudaFuncAttributeMaxDynamicSharedMemorySize, L_SMEM);
     if (e != cudaSuccess) return e;
     const int Kgp = (Kg + 255) & ~255;                   // where the listed components start
     const bool screen = n_listed > 0 && n_slots > 0;
@@ -1570,13 +1770,16 @@ cudaError_t launch_lse_wide(cudaStream_t s, int64_t n, int D, int K, int Kg, int
     LseParams p;
     p.n = n; p.NC = (cols + 127) / 128; p.NZ = atoms;
     p.tkck = reinterpret_cast<const float2*>(wb.tkck); p.cref = wb.cref; p.logz = wb.logz; p.llpart = nullptr; p.status = status;
-    p.top = reinterpret_cast<float4*>(wb.top);
-    p.scr = screen ? reinterpret_cast<const float2*>(wb.scr) : nullptr;
+    p.top = wb.top;
+    p.screen = screen;
+    p.scr = reinterpret_cast<const float2*>(wb.scr);
     p.scr_mask = wb.scr_mask; p.slot_of = wb.slot_of; p.n2 = wb.n2; p.cand = wb.cand;
     p.cand_words = (n_slots + 31) / 32; p.scr_group = Kgp / 256; p.ctl = wb.ctl;
     const int64_t ntiles = (n + WIDE_TILE - 1) / WIDE_TILE;
     const unsigned grid = (unsigned)(ntiles < num_sms ? ntiles : num_sms);
-    lse_wide_kernel<<<grid, WT_THREADS, L_SMEM, s>>>(p, tm_yhi, tm_ylo, tm_phi, tm_plo);
+    if (ntop == 2) lse_wide_kernel<2><<<grid, WT_THREADS, L_SMEM, s>>>(p, tm_yhi, tm_ylo, tm_phi, tm_plo);
+    else if (ntop == 6) lse_wide_kernel<6><<<grid, WT_THREADS, L_SMEM, s>>>(p, tm_yhi, tm_ylo, tm_phi, tm_plo);
+    else lse_wide_kernel<WIDE_MAX_TOP><<<grid, WT_THREADS, L_SMEM, s>>>(p, tm_yhi, tm_ylo, tm_phi, tm_plo);
     return cudaGetLastError();
 }
 

@@ -14,6 +14,7 @@ constexpr int WIDE_BATCH = 256;              // points per batch of the second s
 constexpr int WIDE_TILE = 128;               // points per tile of the first sweep
 constexpr int WIDE_MAX_ILL = 2048;           // ill-conditioned components the FP32 kernels evaluate as a sub-mixture
 constexpr int WIDE_LL_BLOCKS = 64;           // per-block partial sums of the log-likelihood
+constexpr int WIDE_MAX_TOP = 10;             // candidates per point sweep 1 can report (the top-m assignment asks for m + 2)
 constexpr int WIDE_CAND_WORDS = WIDE_MAX_ILL / 32;          // 32-bit words of a point's row of the candidate bitmap
 constexpr int WIDE_CANDT_WORDS = (int)(WIDE_PIECE / 32);    // words of a slot's row of the transposed bitmap
 
@@ -54,11 +55,13 @@ struct WideBuffers {
     unsigned char* y_lo;
     double* logz;   // [WIDE_PIECE] log2 Z of the piece's points as sweep 1 finds it (consistent with sweep 2's logits)
     double* logz_x; // [WIDE_PIECE] the same with the two leading terms of every point replaced by their exact values
-    float* top;     // [WIDE_PIECE][4] per point: its two largest approximate log2 z - c_ref and their components
+    float* top;     // [WIDE_PIECE][2 WIDE_MAX_TOP] per point: its largest approximate log2 z - c_ref, then their positions
+                    // (rows of 2 ntop floats for the ntop of the launch)
     float* partial; // [R * CL][pcols][128] per-CTA partial statistics of the second sweep
     double* llpart; // [WIDE_LL_BLOCKS] partial sums of log Z
     // Screening of the (point, ill-conditioned component) pairs by sweep 1 and their exact evaluation pair by pair:
-    float* scr;     // [rows] pairs: (c - c_ref + error allowance, allowance per unit of |x - g|^2); -inf for the others
+    float* scr;     // [rows] pairs.  Listed components: (c - c_ref + error allowance, allowance per unit of |x - g|^2);
+                    // evaluated components: (error allowance, allowance per unit of |x - g|^2); (-inf, 0) elsewhere
     int* slot_of;   // [rows] slot in the list of the component at a position, -1 if it is not listed
     int* scr_mask;  // [rows / 32] nonzero where a chunk of 32 positions holds a listed component
     float* n2;      // [WIDE_PIECE] |x_i - g|^2
@@ -97,8 +100,15 @@ cudaError_t launch_cand_count_wide(cudaStream_t s, const WideBuffers& wb);
 // n_listed > 0 (listed components, n_slots slots of the list): the sweep also marks in wb.cand every pair of a point and a
 // listed component whose approximate log2 z, raised by its error bound, comes within 2^-40 of the point's maximum, and
 // counts the marks in wb.ctl[0]; wb.n2, wb.cand (zeroed) and wb.ctl (zeroed) must have been prepared for the piece.
+// ntop (2, 6 or WIDE_MAX_TOP): how many of a point's largest approximate values go to wb.top.
 cudaError_t launch_lse_wide(cudaStream_t s, int64_t n, int D, int K, int Kg, int n_listed, int n_slots, const WideBuffers& wb,
-                            int num_sms, int* status);
+                            int num_sms, int* status, int ntop = 2);
+// Top-m assignment of the n points of a piece from what launch_lse_wide (ntop >= m + 2; screened: it also marked the listed
+// pairs) and launch_norm_wide left in wb: idx [n][m], resp [n][m] (may be NULL); rows whose answer is not certain are appended to unc_rows
+// (unc_count += 1 each) and left unwritten.  mu, w2, c2d: the FP32 path's derived parameters.
+cudaError_t launch_assign_refine_wide(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu, const float* w2,
+                                      const double* c2d, int n_slots, bool screened, const WideBuffers& wb, int ntop, int m,
+                                      int32_t* idx, float* resp, int32_t* unc_rows, int* unc_count, bool index_only);
 // wb.n2[i] = |x_i - g|^2 for the n points of a piece.
 cudaError_t launch_norm_wide(cudaStream_t s, const float* X, int64_t n, int D, const WideBuffers& wb);
 // Clears wb.ctl, the n rows of wb.cand and the n_slots rows of wb.candT before a piece's first sweep.

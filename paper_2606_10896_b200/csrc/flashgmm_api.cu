@@ -116,7 +116,7 @@ ScratchLayout scratch_layout(int D, int K, bool planes) {
         L.w_candT = take((size_t)WIDE_MAX_ILL * WIDE_CANDT_WORDS * 4);
         L.w_ctl = take(32);
         L.w_logz = take((size_t)WIDE_PIECE * 8);
-        L.w_top = take((size_t)WIDE_PIECE * 16);
+        L.w_top = take((size_t)WIDE_PIECE * 2 * WIDE_MAX_TOP * 4);
         L.w_logzx = take((size_t)WIDE_PIECE * 8);
         L.w_partial_bytes = (size_t)wp.R * wp.CL * wp.pcols * 128 * 4;
         L.w_partial = take(L.w_partial_bytes);
@@ -949,6 +949,65 @@ int assign_topm_impl(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, cons
     // exactly for every point; parameters with more than TC_MAX_ILL of them (a flag written on the device by the
     // preparation kernels) go through the FP32 kernels instead: both sets of kernels are enqueued and each checks the
     // flag, so the call stays asynchronous.
+    if (wide_supports(D, K)) {
+        // Wide data: the first sweep of the two-sweep tensor path reports every point's m + 2 largest approximate values and
+        // marks the listed (ill-conditioned) components that can matter; a warp per point then evaluates those exactly.  Rows
+        // whose answer is not certain, pieces with too many marked pairs, and parameter sets with too many listed components
+        // go through the FP32 kernels.
+        const bool want = ctx->capPlanes && ctx->lay.wide && ctx->path != GMM_PATH_FP32 && K >= 64 && m + 2 <= WIDE_MAX_TOP;
+        bool tensor_w = false;
+        if (want) {
+            const WideBuffers wb = ctx->wide();
+            const float limit = ctx->tc_cond_limit >= 0.f ? ctx->tc_cond_limit : 0.01f;
+            KL(launch_prepare_wide(ctx->stream, D, K, pi, mu, var, wb, limit, 0.f));
+            ctx->launches += 4;
+            int fl[8];
+            CU(cudaMemcpyAsync(fl, wb.flags, sizeof(fl), cudaMemcpyDeviceToHost, ctx->stream));
+            CU(cudaStreamSynchronize(ctx->stream));
+            const int n_ill = fl[4], Kg = fl[6], n_list = fl[2];
+            if (n_ill + 64 <= WIDE_MAX_ILL && 2 * n_ill <= K && Kg >= 1) {
+                tensor_w = true;
+                if (n_ill > 0) KL(launch_ill_gather_wide(ctx->stream, D, n_list, wb, mu, ctx->w2(), ctx->c2d()));
+                // (ten reported candidates instead of six for m <= 4 leave no fewer rows to the FP32 kernels: the rows that
+                // go there have broad posteriors, with more than ten components above 1e-3 of Z between them)
+                const int ntop = (m + 2 <= 6) ? 6 : WIDE_MAX_TOP;
+                const bool screen = n_ill > 0;
+                const int64_t piece = ctx->wide_piece;
+                const int64_t cap = N < piece ? N : piece;
+                const size_t need = align256((size_t)cap * sizeof(int32_t)) + 256;       // uncertain rows of a piece, their count
+                CHECK(grow_buffer(ctx, &ctx->at_scratch, &ctx->at_scratch_bytes, need, "the assignment's list of uncertain rows"));
+                unsigned char* base = static_cast<unsigned char*>(ctx->at_scratch);
+                int32_t* unc_rows = reinterpret_cast<int32_t*>(base);
+                int* unc_count = reinterpret_cast<int*>(base + need - 256);
+                for (int64_t off = 0; off < N; off += piece) {
+                    const int64_t cnt = (N - off < piece) ? (N - off) : piece;
+                    const float* Xs = X + off * D;
+                    int32_t* idx_p = idx + off * m;
+                    float* resp_p = resp ? resp + off * m : nullptr;
+                    CU(cudaMemsetAsync(unc_count, 0, sizeof(int), ctx->stream));
+                    if (screen) CU(launch_cand_clear_wide(ctx->stream, cnt, n_list, wb));
+                    CHECK(prof_begin(ctx));
+                    KL(launch_norm_wide(ctx->stream, Xs, cnt, D, wb));
+                    KL(launch_transform_wide(ctx->stream, Xs, cnt, D, wb, &ctx->result()->status));
+                    KL(launch_lse_wide(ctx->stream, cnt, D, K, Kg, screen ? n_ill : 0, n_list, wb, ctx->sms, &ctx->result()->status, ntop));
+                    if (screen) KL(launch_cand_gate_wide(ctx->stream, wb, ctx->wide_sparse >= 2 ? ((long long)1 << 62) : (long long)cnt * n_list / 64));
+                    KL(launch_assign_refine_wide(ctx->stream, Xs, cnt, D, K, mu, ctx->w2(), ctx->c2d(), n_list, screen, wb, ntop, m, idx_p, resp_p,
+                                                 unc_rows, unc_count, index_only));
+                    // the rows left uncertain, against all K components; and the whole piece if its marked pairs were too many
+                    KL(launch_topm_fp32(ctx->stream, Xs, cnt, D, K, mu, ctx->w2(), ctx->c2d(), ctx->center(), m, idx_p, resp_p, nullptr, unc_rows, unc_count));
+                    if (screen) KL(launch_topm_fp32(ctx->stream, Xs, cnt, D, K, mu, ctx->w2(), ctx->c2d(), ctx->center(), m, idx_p, resp_p, wb.ctl + 1));
+                    CHECK(prof_end(ctx));
+                }
+            }
+        }
+        if (!tensor_w)
+            for (int64_t off = 0; off < N; off += SUPER_TILE) {
+                const int64_t cnt = (N - off < SUPER_TILE) ? (N - off) : SUPER_TILE;
+                KL(launch_topm_fp32(ctx->stream, X + off * D, cnt, D, K, mu, ctx->w2(), ctx->c2d(), ctx->center(), m, idx + off * m, resp ? resp + off * m : nullptr, nullptr));
+            }
+        ctx->last_path = tensor_w ? GMM_PATH_TENSOR : GMM_PATH_FP32;
+        return GMM_OK;
+    }
     const bool tensor = ctx->capPlanes && ctx->lay.tc && ctx->path != GMM_PATH_FP32;
     const int* run_fp32_if = nullptr;
     if (tensor) {

@@ -12,15 +12,23 @@ Tolerance of the GPU comparison, per coordinate (k, d) of a group of T points, w
 group's share N_k / T of component k over the square root of the component's weight (about sqrt(pi_k) <= 1 for a group
 that resembles the mixture, up to 1 / sqrt(pi_k) for a group that sits on one light component):
 
-    2e-5 (1 + max|G|)  +  A_k (0.5 e + 4e-5 (1 + mu_kd^2 / var_kd))
+    f x [ 2e-5 (1 + max|G|)  +  A_k (0.5 e + 4e-5 (1 + mu_kd^2 / var_kd)) ]
 
-First term: rounding of the statistics for ordinary coordinates.  Last term: a coordinate is a difference of the raw
-moments N_k, S1, S2, which the tile kernels deliver to about 4e-6 relative (tensor path; 2e-7 on the FP32 path), and the
-difference cancels by (1 + mu^2 / var).  Middle term: an error e (in bits) of a logit moves a contested responsibility by
-up to r (1 - r) ln 2 e <= 0.17 e, coherently over points that share a region, and enters a coordinate times |z| or
-|z^2 - 1| (taken as 3).  On the tensor path e = 8 x 1.5e-4 sqrt(N / K) bits, the kernel's own error bound for the
-components it does not recompute exactly (N = all points of the call); on the FP32 path e = 2e-4 bits (fp32 rounding
-of logits of a few hundred bits).
+The bracket is a worst-case bound.  First term: rounding of the statistics for ordinary coordinates.  Last term: a
+coordinate is a difference of the raw moments N_k, S1, S2, which the tile kernels deliver to about 4e-6 relative (tensor
+path; 2e-7 on the FP32 path), and the difference cancels by (1 + mu^2 / var).  Middle term: an error e (in bits) of a
+logit moves a contested responsibility by up to r (1 - r) ln 2 e <= 0.17 e, coherently over points that share a region,
+and enters a coordinate times |z| or |z^2 - 1| (taken as 3).  On the tensor path e = 8 x 1.5e-4 sqrt(N / K) bits, the
+kernel's own error bound for the components it does not recompute exactly (N = all points of the call); on the FP32
+path e = 2e-4 bits (fp32 rounding of logits of a few hundred bits).
+
+The factor f brings the bound down to about ten times the error measured in each regime (largest |dG| / bracket over
+this file's cases, B200):
+    groups drawn from the mixture (every test but the one below), either path:   0.013 measured,  f = 0.1
+    a group that sits on one light component next to a close copy of it (the bound's worst case: every responsibility
+    of the group contested, A_k near 1 / (2 sqrt(pi_k)) = 50):
+        tensor path   0.084 (K = 256, D = 64) and 0.31 (K = 1024, D = 128) measured,   f = 1
+        FP32 path     0.0013 and 0.0040 measured,                                     f = 0.04
 """
 import numpy as np
 import pytest
@@ -167,8 +175,9 @@ def _run_gpu(X, offsets, pi, mu, var, path=None, repeat=True):
     return fv.cpu().numpy().astype(np.float64), ll, used
 
 
-def _tolerance(G_ref, X, offsets, pi, mu, var, tensor_path):
+def _tolerance(G_ref, X, offsets, pi, mu, var, tensor_path, contested=False):
     """The per-coordinate bound of this file's header."""
+    f = (1.0 if tensor_path else 0.04) if contested else 0.1
     n_all = int(sum(int(offsets[g + 1]) - int(offsets[g]) for g in range(len(offsets) - 1)))
     e_bits = 8 * 1.5e-4 * np.sqrt(max(n_all, 1) / len(pi)) if tensor_path else 2e-4
     tol = np.full(G_ref.shape, 2e-5 * (1.0 + np.abs(G_ref).max()))
@@ -181,17 +190,17 @@ def _tolerance(G_ref, X, offsets, pi, mu, var, tensor_path):
         Nk = gmm_oracle.em_step(X[lo:hi], pi, mu, var)[0]
         A = np.where(pi64 > 0, Nk / ((hi - lo) * np.sqrt(np.where(pi64 > 0, pi64, 1.0))), 0.0)
         tol[g] += (A[:, None] * (0.5 * e_bits + 4e-5 * ratio))[None]
-    return tol
+    return f * tol
 
 
-def _check_against_oracle(X, offsets, pi, mu, var, path=None):
+def _check_against_oracle(X, offsets, pi, mu, var, path=None, contested=False):
     G_ref = fisher_vectors(X, offsets, pi, mu, var)
     lo, hi = int(offsets[0]), int(offsets[-1])
     ll_ref = float(gmm_oracle.responsibilities(X[lo:hi], pi, mu, var)[1].sum()) if hi > lo else 0.0
     G_gpu, ll, used = _run_gpu(X, offsets, pi, mu, var, path)
     assert G_gpu.shape == G_ref.shape and np.isfinite(G_gpu).all()
     from paper_2606_10896_b200 import flashgmm as fg
-    tol = _tolerance(G_ref, X, offsets, pi, mu, var, used == fg.GMM_PATH_TENSOR)
+    tol = _tolerance(G_ref, X, offsets, pi, mu, var, used == fg.GMM_PATH_TENSOR, contested)
     excess = np.abs(G_gpu - G_ref) - tol
     worst = np.unravel_index(np.argmax(excess), excess.shape)
     assert excess.max() <= 0, f"|dG| = {np.abs(G_gpu - G_ref)[worst]:.3e} > {tol[worst]:.3e} at (group, part, k, d) = {worst}"
@@ -267,7 +276,7 @@ def test_gpu_fisher_vectors_of_a_group_that_sits_on_one_light_component(K, D, T)
     X = np.concatenate(parts)
     offsets = np.array([0, T, 2 * T, 2 * T + T // 2], np.int64)
     for path in (fg.GMM_PATH_TENSOR, fg.GMM_PATH_FP32):
-        _check_against_oracle(X, offsets, pi, mu, var, path)
+        _check_against_oracle(X, offsets, pi, mu, var, path, contested=True)
 
 
 @pytest.mark.gpu

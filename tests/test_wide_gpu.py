@@ -215,3 +215,71 @@ def test_many_marked_pairs_go_to_the_dense_kernels(fg, ctx):
     _step_and_check(fg, ctx, X, pi, mu, var, "overlapping clusters, light components")
     marked, kept, dense = ctx.gmm_last_exact_pairs()
     assert ctx.gmm_last_exact_count() >= 6 and dense == 1 and marked > 24_000 * 6 // 64
+
+
+# ---- top-m assignment on wide data (paper Sections 4.2-4.3) ---------------------------------------------------------
+
+def _assign_and_check(fg, ctx, X, pi, mu, var, m, what, indices_only=False):
+    from tests.parity_util import assert_topm_matches, oracle_resp_at
+
+    idx, resp = ctx.gmm_assign_topm(_t(X), _t(pi), _t(mu), _t(var), m, indices_only=indices_only)
+    ctx.gmm_sync_status()
+    idx_g = idx.cpu().numpy()
+    resp_g = None if resp is None else resp.cpu().numpy()
+    idx_r, resp_r, next_r = orc.topm(X, pi, mu, var, m)
+    assert idx_g.min() >= 0 and idx_g.max() < len(pi), f"{what}: index out of range"
+    for row in idx_g[:: max(1, len(idx_g) // 500)]:
+        assert len(set(row.tolist())) == m, f"{what}: repeated component in a row"
+    r_at_g = oracle_resp_at(orc, X, pi, mu, var, idx_g)
+    assert_topm_matches(idx_g, resp_g, idx_r, resp_r, next_r, r_at_g, what=what, check_values=resp_g is not None)
+    return idx_g, resp_g
+
+
+@pytest.mark.parametrize("m", [1, 2, 4, 8])
+def test_wide_assignment_against_oracle(fg, ctx, m):
+    """Tiles with a ragged tail, a ragged last slice of dimensions and of components; m + 2 <= 6 and m + 2 = 10 reported
+    candidates."""
+    X, pi, mu, var = _clustered(np.random.default_rng(100 + m), 9_000 + 77, 200, 130)
+    ctx.gmm_set_path(fg.GMM_PATH_TENSOR)
+    _assign_and_check(fg, ctx, X, pi, mu, var, m, f"wide assignment m={m}")
+    assert ctx.gmm_last_path() == fg.GMM_PATH_TENSOR
+    if m == 4:
+        _assign_and_check(fg, ctx, X, pi, mu, var, m, "wide assignment, indices only", indices_only=True)
+
+
+def test_wide_assignment_with_listed_components_ties_and_overlap(fg, monkeypatch):
+    """(a) Collapsed components own their point; (b) two identical components tie exactly on every point of their cluster
+    (the smaller index first); (c) clusters that overlap: many components matter for a point, the rows go to the FP32
+    kernels; (d) pieces of 4096 points."""
+    monkeypatch.setenv("GMM_WIDE_PIECE", "4096")
+    rng = np.random.default_rng(55)
+    X, pi, mu, var = _with_listed_components(rng, 12_000, 288, 80)
+    mu[40], var[40], pi[40] = mu[41], var[41], pi[41]          # an exact copy: ties
+    pi = (pi / pi.sum()).astype(np.float32)
+    with fg.Context(0) as c:
+        c.gmm_set_path(fg.GMM_PATH_TENSOR)
+        idx, resp = _assign_and_check(fg, c, X, pi, mu, var, 4, "wide assignment with listed components")
+        assert c.gmm_last_path() == fg.GMM_PATH_TENSOR
+        for j in range(5):                                      # the point a collapsed component sits on
+            assert idx[50 + j, 0] == j and resp[50 + j, 0] > 0.999
+        tied = np.flatnonzero((idx[:, 0] == 40) | (idx[:, 0] == 41))
+        assert len(tied) > 50 and np.all(idx[tied, 0] == 40) and np.all(idx[tied, 1] == 41)
+        Xo, pio, muo, varo = _clustered(np.random.default_rng(56), 6_000, 256, 64, sep=0.02)
+        _assign_and_check(fg, c, Xo, pio, muo, varo, 4, "wide assignment, overlapping clusters")
+
+
+def test_wide_assignment_path_choice(fg, ctx):
+    """AUTO takes the tensor path for K >= 64; FP32 when forced, for small K, or when more than half of the components are
+    ill-conditioned."""
+    X, pi, mu, var = _clustered(np.random.default_rng(8), 5_000, 256, 64)
+    ctx.gmm_set_path(fg.GMM_PATH_AUTO)
+    _assign_and_check(fg, ctx, X, pi, mu, var, 2, "AUTO")
+    assert ctx.gmm_last_path() == fg.GMM_PATH_TENSOR
+    ctx.gmm_set_path(fg.GMM_PATH_FP32)
+    _assign_and_check(fg, ctx, X, pi, mu, var, 2, "FP32 forced")
+    assert ctx.gmm_last_path() == fg.GMM_PATH_FP32
+    ctx.gmm_set_path(fg.GMM_PATH_AUTO)
+    v2 = var.copy()
+    v2[:40] = 1e-6
+    _assign_and_check(fg, ctx, X, pi, mu, v2, 2, "40 of 64 collapsed")
+    assert ctx.gmm_last_path() == fg.GMM_PATH_FP32

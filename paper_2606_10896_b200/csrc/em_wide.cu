@@ -294,7 +294,8 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
         // Item order = order of use: per (tile, group, atom z) the tile's Y atom, then the group's coefficient atoms.
         int64_t g = 0;
         bool ok = true;
-        auto item = [&](const CUtensorMap* mh, const CUtensorMap* ml, int32_t row, int32_t z) -> bool {
+        const uint64_t pol_keep = l2_policy_evict_last(), pol_stream = l2_policy_evict_first();
+        auto item = [&](const CUtensorMap* mh, const CUtensorMap* ml, int32_t row, int32_t z, bool keep) -> bool {
             const int slot = (int)(g % L_SLOTS);
             const int64_t use = g / L_SLOTS;
             if (use > 0) {
@@ -305,8 +306,9 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
             if (elect_one()) {
                 const uint32_t dst = smem_u32(smem + slot * SLOT);
                 bar_expect_tx(BAR(LB_FULL + slot), SLOT);
-                tma_load_3d(dst, mh, 0, row, z, BAR(LB_FULL + slot));
-                tma_load_3d(dst + SLOT / 2, ml, 0, row, z, BAR(LB_FULL + slot));
+                // the coefficient atoms are read by every CTA for every tile, the tile's own atoms once
+                tma_load_3d_hint(dst, mh, 0, row, z, BAR(LB_FULL + slot), keep ? pol_keep : pol_stream);
+                tma_load_3d_hint(dst + SLOT / 2, ml, 0, row, z, BAR(LB_FULL + slot), keep ? pol_keep : pol_stream);
             }
             __syncwarp();
             ++g;
@@ -317,8 +319,8 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
             for (int gq = 0; gq < NG && ok; ++gq) {
                 const int nch = (NC - 2 * gq < 2) ? (NC - 2 * gq) : 2;
                 for (int z = 0; z < NZ && ok; ++z) {
-                    ok = item(&tm_yhi, &tm_ylo, row0, z);
-                    for (int c = 0; c < nch && ok; ++c) ok = item(&tm_phi, &tm_plo, (2 * gq + c) * 128, z);
+                    ok = item(&tm_yhi, &tm_ylo, row0, z, false);
+                    for (int c = 0; c < nch && ok; ++c) ok = item(&tm_phi, &tm_plo, (2 * gq + c) * 128, z, true);
                 }
             }
         }
@@ -547,6 +549,7 @@ em_wide_kernel(const EmWideParams p, const __grid_constant__ CUtensorMap tm_phi,
         // batch: 64 points x 2 atoms of both planes (2 x 16 KB in one slot).
         int64_t g = 0;
         bool ok = true;
+        const uint64_t pol_keep = l2_policy_evict_last();     // the slice's coefficient atoms come back with every batch
         auto acquire = [&]() -> int {
             const int slot = (int)(g % E_SLOTS);
             const int64_t use = g / E_SLOTS;
@@ -565,8 +568,8 @@ em_wide_kernel(const EmWideParams p, const __grid_constant__ CUtensorMap tm_phi,
                 if (elect_one()) {
                     const uint32_t dst = smem_u32(smem + slot * SLOT);
                     bar_expect_tx(BAR(EB_FULL + slot), SLOT);
-                    tma_load_3d(dst, &tm_phi, 0, slice * 128, z, BAR(EB_FULL + slot));
-                    tma_load_3d(dst + SLOT / 2, &tm_plo, 0, slice * 128, z, BAR(EB_FULL + slot));
+                    tma_load_3d_hint(dst, &tm_phi, 0, slice * 128, z, BAR(EB_FULL + slot), pol_keep);
+                    tma_load_3d_hint(dst + SLOT / 2, &tm_plo, 0, slice * 128, z, BAR(EB_FULL + slot), pol_keep);
                 }
                 __syncwarp();
                 ++g;
@@ -707,9 +710,11 @@ em_wide_kernel(const EmWideParams p, const __grid_constant__ CUtensorMap tm_phi,
 }
 
 // ------------------------------------------------------------------------------------------------------------------
-// X -> the two fp16 planes of Y = [u | u^2 + kap], u = s_d (x - g_d).  Row i of a plane holds 2 Dpad halves: k-step ks (8
-// dimensions) occupies halves [16 ks, 16 ks + 8) = u and [16 ks + 8, 16 ks + 16) = u^2 + kap.  One thread converts one
-// (point, k-step) unit and writes 32 contiguous bytes per plane.  Rows n .. rows_padded - 1 are written as zeros.
+// X -> the two fp16 planes of Y = [u | u^2 + kap], u = s_d (x - g_d).  A point has 2 Dpad halves per plane: k-step ks (8
+// dimensions) occupies halves [16 ks, 16 ks + 8) = u and [16 ks + 8, 16 ks + 16) = u^2 + kap.  A plane is stored atom by
+// atom (an atom = 64 halves = 4 k-steps of every point: [atom][point][128 bytes]), so that the tiles the sweeps load -
+// some rows of one atom - are contiguous in memory.  One thread converts one (point, k-step) unit and writes 32
+// contiguous bytes per plane.  Rows n .. rows_padded - 1 are written as zeros.
 __global__ void __launch_bounds__(256) wide_transform_kernel(const float* __restrict__ X, int64_t n, int64_t rows_padded, int D,
                                                              int Dpad, const float* __restrict__ sd, const float* __restrict__ kap,
                                                              const float* __restrict__ gd, unsigned char* __restrict__ yhi,
@@ -718,7 +723,6 @@ __global__ void __launch_bounds__(256) wide_transform_kernel(const float* __rest
     const int64_t units = rows_padded * upr;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     const bool vec_ok = (D % 4 == 0) && ((reinterpret_cast<uintptr_t>(X) & 15) == 0);
-    const size_t pitch = (size_t)Dpad * 4;               // bytes per row of a plane
     bool bad = false;
     for (int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; u < units; u += stride) {
         const int64_t row = u / upr;
@@ -755,8 +759,9 @@ __global__ void __launch_bounds__(256) wide_transform_kernel(const float* __rest
             qh[j / 2] = *reinterpret_cast<const uint32_t*>(&sq);
             ql[j / 2] = *reinterpret_cast<const uint32_t*>(&t2);
         }
-        uint4* oh = reinterpret_cast<uint4*>(yhi + row * pitch + ks * 32);
-        uint4* ol = reinterpret_cast<uint4*>(ylo + row * pitch + ks * 32);
+        const size_t o = ((size_t)(ks >> 2) * rows_padded + row) * 128 + (ks & 3) * 32;      // [atom][row][128 bytes]
+        uint4* oh = reinterpret_cast<uint4*>(yhi + o);
+        uint4* ol = reinterpret_cast<uint4*>(ylo + o);
         oh[0] = make_uint4(xh[0], xh[1], xh[2], xh[3]);
         oh[1] = make_uint4(qh[0], qh[1], qh[2], qh[3]);
         ol[0] = make_uint4(xl[0], xl[1], xl[2], xl[3]);
@@ -990,7 +995,7 @@ __global__ void __launch_bounds__(1024) wide_ill_list_kernel(int K, int rows, co
 
 // One block per position of the tensor passes: coefficient planes, t, c (float64) of the component that sits there
 // (zero planes and c = -inf for an empty position).
-__global__ void __launch_bounds__(256) wide_prepare_kernel(int D, int Dpad, const int* __restrict__ comp_of, const float* __restrict__ pi,
+__global__ void __launch_bounds__(256) wide_prepare_kernel(int D, int Dpad, int rows, const int* __restrict__ comp_of, const float* __restrict__ pi,
                                                            const float* __restrict__ mu, const float* __restrict__ var,
                                                            const float* __restrict__ sd, const float* __restrict__ kap,
                                                            const float* __restrict__ gd, __half* __restrict__ p_hi,
@@ -1027,14 +1032,14 @@ __global__ void __launch_bounds__(256) wide_prepare_kernel(int D, int Dpad, cons
     double tt = 1.0;
     if (mx > 0.0 && isfinite(mx)) tt = exp2(floor(log2(mx)) - 9.0);      // max |P / t| in [512, 1024)
     double ksum = 0.0;
-    __half* rh = p_hi + (size_t)pos * 2 * Dpad;
-    __half* rl = p_lo + (size_t)pos * 2 * Dpad;
+    // planes stored atom by atom: [atom of 64 columns][position][64 halves]
+    auto at = [&](int cx) { return ((size_t)(cx >> 6) * rows + pos) * 64 + (cx & 63); };
     for (int d = t; d < Dpad; d += 256) {
         const double as = ab_s[d] / tt, bs = ab_s[Dpad + d] / tt;
         const __half ah = __double2half(as), bh = __double2half(bs);
         const __half al = __double2half(as - (double)__half2float(ah)), bl = __double2half(bs - (double)__half2float(bh));
         const int cx = 16 * (d >> 3) + (d & 7);          // k-step interleaved column order, slices of 128 dimensions in sequence
-        rh[cx] = ah; rh[cx + 8] = bh; rl[cx] = al; rl[cx + 8] = bl;
+        p_hi[at(cx)] = ah; p_hi[at(cx + 8)] = bh; p_lo[at(cx)] = al; p_lo[at(cx + 8)] = bl;
         // what the contraction adds through the shifted squares is taken out of c_k; so is what the rounding of the
         // coefficients (22 bits of the row's largest entry: the same error for every point) makes it miss at the
         // component's own mean u = s (mu - g), which leaves an error proportional to a point's distance from that mean
@@ -1582,11 +1587,12 @@ __global__ void wide_ill_scatter_kernel(int D, int K, int n_ill, const int* __re
     }
 }
 
-// A plane [rows][pitch bytes] seen as a 3-D tensor (x = 64 halves of an atom's row, y = row, z = atom): a box of
-// (64, box_rows, box_atoms) lands in shared memory as [atom][row][128 bytes], each 128-byte row swizzled.
-cudaError_t wide_make_map(CUtensorMap* tm, void* base, int64_t rows, int64_t pitch, int atoms, int box_rows, int box_atoms) {
+// A plane [atoms][rows][128 bytes] seen as a 3-D tensor (x = 64 halves of an atom's row, y = row, z = atom): a box of
+// (64, box_rows, box_atoms) is box_atoms contiguous blocks of box_rows x 128 bytes in memory and lands in shared memory as
+// [atom][row][128 bytes], each 128-byte row swizzled.
+cudaError_t wide_make_map(CUtensorMap* tm, void* base, int64_t rows, int atoms, int box_rows, int box_atoms) {
     const cuuint64_t dims[3] = {64, (cuuint64_t)rows, (cuuint64_t)atoms};
-    const cuuint64_t strides[2] = {(cuuint64_t)pitch, 128};
+    const cuuint64_t strides[2] = {128, (cuuint64_t)rows * 128};
     const cuuint32_t box[3] = {64, (cuuint32_t)box_rows, (cuuint32_t)box_atoms};
     const cuuint32_t estr[3] = {1, 1, 1};
     typedef CUresult (*encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -1642,7 +1648,7 @@ cudaError_t launch_prepare_wide(cudaStream_t s, int D, int K, const float* pi, c
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     wide_prepare_kernel<<<pl.rows, 256, (size_t)2 * pl.Dpad * sizeof(double), s>>>(
-        D, pl.Dpad, wb.comp_of, pi, mu, var, wb.sd, wb.kap, wb.gd, reinterpret_cast<__half*>(wb.p_hi),
+        D, pl.Dpad, pl.rows, wb.comp_of, pi, mu, var, wb.sd, wb.kap, wb.gd, reinterpret_cast<__half*>(wb.p_hi),
         reinterpret_cast<__half*>(wb.p_lo), wb.tk, wb.ckd);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
@@ -1750,13 +1756,12 @@ cudaError_t launch_lse_wide(cudaStream_t s, int64_t n, int D, int K, int Kg, int
     if (n < 1 || n > WIDE_PIECE || Kg < 1 || Kg > K) return cudaErrorInvalidValue;
     const WidePlan pl = wide_plan(D, K, num_sms);
     const int64_t rp = rows_padded_of(n);
-    const int64_t pitch = (int64_t)pl.Dpad * 4;
     const int atoms = 4 * pl.n_slices;
     CUtensorMap tm_yhi, tm_ylo, tm_phi, tm_plo;
-    cudaError_t e = wide_make_map(&tm_yhi, wb.y_hi, rp, pitch, atoms, WIDE_TILE, 1);
-    if (e == cudaSuccess) e = wide_make_map(&tm_ylo, wb.y_lo, rp, pitch, atoms, WIDE_TILE, 1);
-    if (e == cudaSuccess) e = wide_make_map(&tm_phi, wb.p_hi, pl.rows, pitch, atoms, 128, 1);
-    if (e == cudaSuccess) e = wide_make_map(&tm_plo, wb.p_lo, pl.rows, pitch, atoms, 128, 1);
+    cudaError_t e = wide_make_map(&tm_yhi, wb.y_hi, rp, atoms, WIDE_TILE, 1);
+    if (e == cudaSuccess) e = wide_make_map(&tm_ylo, wb.y_lo, rp, atoms, WIDE_TILE, 1);
+    if (e == cudaSuccess) e = wide_make_map(&tm_phi, wb.p_hi, pl.rows, atoms, 128, 1);
+    if (e == cudaSuccess) e = wide_make_map(&tm_plo, wb.p_lo, pl.rows, atoms, 128, 1);
     if (ntop != 2 && ntop != 6 && ntop != WIDE_MAX_TOP) return cudaErrorInvalidValue;
     if (e == cudaSuccess)
         e = ntop == 2 ? cudaFuncSetAttribute(lse_wide_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, L_SMEM)
@@ -1788,15 +1793,14 @@ cudaError_t launch_em_wide(cudaStream_t s, int64_t n, int D, int K, int Kg, cons
     const WidePlan pk = wide_plan(D, K, num_sms);
     const WidePlan pl = wide_plan(D, Kg, num_sms);       // the sweep covers the evaluated positions only
     const int64_t rp = rows_padded_of(n);
-    const int64_t pitch = (int64_t)pl.Dpad * 4;
     const int atoms = 4 * pl.n_slices;
     CUtensorMap tm_phi, tm_plo, tm_ye_hi, tm_ye_lo, tm_ym_hi, tm_ym_lo;
-    cudaError_t e = wide_make_map(&tm_phi, wb.p_hi, pk.rows, pitch, atoms, 128, 1);
-    if (e == cudaSuccess) e = wide_make_map(&tm_plo, wb.p_lo, pk.rows, pitch, atoms, 128, 1);
-    if (e == cudaSuccess) e = wide_make_map(&tm_ye_hi, wb.y_hi, rp, pitch, atoms, WIDE_BATCH, 1);
-    if (e == cudaSuccess) e = wide_make_map(&tm_ye_lo, wb.y_lo, rp, pitch, atoms, WIDE_BATCH, 1);
-    if (e == cudaSuccess) e = wide_make_map(&tm_ym_hi, wb.y_hi, rp, pitch, atoms, 64, 2);
-    if (e == cudaSuccess) e = wide_make_map(&tm_ym_lo, wb.y_lo, rp, pitch, atoms, 64, 2);
+    cudaError_t e = wide_make_map(&tm_phi, wb.p_hi, pk.rows, atoms, 128, 1);
+    if (e == cudaSuccess) e = wide_make_map(&tm_plo, wb.p_lo, pk.rows, atoms, 128, 1);
+    if (e == cudaSuccess) e = wide_make_map(&tm_ye_hi, wb.y_hi, rp, atoms, WIDE_BATCH, 1);
+    if (e == cudaSuccess) e = wide_make_map(&tm_ye_lo, wb.y_lo, rp, atoms, WIDE_BATCH, 1);
+    if (e == cudaSuccess) e = wide_make_map(&tm_ym_hi, wb.y_hi, rp, atoms, 64, 2);
+    if (e == cudaSuccess) e = wide_make_map(&tm_ym_lo, wb.y_lo, rp, atoms, 64, 2);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(em_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, E_SMEM);
     if (e != cudaSuccess) return e;
     EmWideParams p;

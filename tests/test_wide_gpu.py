@@ -283,3 +283,51 @@ def test_wide_assignment_path_choice(fg, ctx):
     v2[:40] = 1e-6
     _assign_and_check(fg, ctx, X, pi, mu, v2, 2, "40 of 64 collapsed")
     assert ctx.gmm_last_path() == fg.GMM_PATH_FP32
+
+
+def test_wide_path_at_its_largest_shape(fg, ctx):
+    """D = 1024 and K = 4096, the limits of the path, on 560,000 device-generated points (just above the 128 points per
+    component from which AUTO takes it).  No oracle step of this size is affordable: the tensor path against the FP32 kernels
+    over the same rows at the ordinary tolerances (the FP32 kernels are checked against the oracle at this D in the cases
+    above), conservation of the weights, and the top-4 assignment against the oracle on a subsample of 1,500 rows."""
+    N, D, K = 560_000, 1024, 4096
+    g = torch.Generator(device=DEV)
+    g.manual_seed(20260611)
+    centres = torch.randn(K, D, device=DEV, generator=g) * 0.3
+    z = torch.randint(0, K, (N,), device=DEV, generator=g)
+    X = centres[z]
+    X += 0.3 * torch.randn(N, D, device=DEV, generator=g)
+    X = X.contiguous()
+    del z
+    pi = np.full(K, 1.0 / K, np.float32)
+    mu = (centres + 0.015 * torch.randn(K, D, device=DEV, generator=g)).cpu().numpy()
+    var = (0.09 * (0.8 + 0.45 * torch.rand(K, D, device=DEV, generator=g))).cpu().numpy()
+    s = float(np.sqrt(X[:50_000].double().var(0).mean().item()))
+    ctx.gmm_set_path(fg.GMM_PATH_AUTO)
+    Nk, S1, S2, L = ctx.gmm_em_step(X, _t(pi), _t(mu), _t(var))
+    assert ctx.gmm_last_path() == fg.GMM_PATH_TENSOR
+    t_ = (Nk.cpu().numpy(), S1.cpu().numpy(), S2.cpu().numpy(), L)
+    assert abs(t_[0].sum() - N) <= 1e-5 * N
+    ctx.gmm_set_path(fg.GMM_PATH_FP32)
+    Nk, S1, S2, Lf = ctx.gmm_em_step(X, _t(pi), _t(mu), _t(var))
+    f_ = (Nk.cpu().numpy(), S1.cpu().numpy(), S2.cpu().numpy(), Lf)
+    what = "D = 1024, K = 4096: tensor vs FP32 path"
+    assert abs(t_[3] - f_[3]) <= 1e-5 * abs(f_[3]), what
+    assert_stats_close(N, s, t_[:3], f_[:3], what)
+
+    def params(st):
+        pi_d, mu_d, var_d = _t(pi), _t(mu), _t(var)
+        ctx.gmm_finalize(N, _t(st[0], torch.float64), _t(st[1], torch.float64), _t(st[2], torch.float64), 1e-6, pi_d, mu_d, var_d)
+        return pi_d.cpu().numpy(), mu_d.cpu().numpy(), var_d.cpu().numpy()
+
+    assert_params_close(N, s, params(t_), params(f_), f_[0], what)
+    ctx.gmm_set_path(fg.GMM_PATH_AUTO)
+    idx, resp = ctx.gmm_assign_topm(X, _t(pi), _t(mu), _t(var), 4)
+    ctx.gmm_sync_status()
+    assert ctx.gmm_last_path() == fg.GMM_PATH_TENSOR
+    rows = torch.as_tensor(synth.subsample_rows(N, 1500, 7), device=DEV)
+    Xs = X[rows].cpu().numpy()
+    from tests.parity_util import assert_topm_matches, oracle_resp_at
+    idx_g, resp_g = idx[rows].cpu().numpy(), resp[rows].cpu().numpy()
+    idx_r, resp_r, next_r = orc.topm(Xs, pi, mu, var, 4)
+    assert_topm_matches(idx_g, resp_g, idx_r, resp_r, next_r, oracle_resp_at(orc, Xs, pi, mu, var, idx_g), what="largest shape, top-4")

@@ -66,6 +66,7 @@ struct LseParams {
     bool screen;         // listed components follow the evaluated ones and are screened
     const float2* scr;   // [NC * 128] listed components: (c - c_ref + error allowance, allowance per unit of |x - g|^2);
                          // evaluated components: (error allowance, allowance per unit of |x - g|^2)
+    const float* scr_e;  // [NC * 128] listed components: the error allowance alone
     const int* scr_mask; // [NC * 4] nonzero where a chunk of 32 components holds a listed one
     const int* slot_of;  // [NC * 128]
     const float* n2;     // [n]
@@ -160,10 +161,21 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
             for (int g = 0; g < NG; ++g) {
                 const int nch = (NC - 2 * g < 2) ? (NC - 2 * g) : 2;
                 const bool screening = p.screen && g >= p.scr_group;
-                if (screening && g == p.scr_group) {          // the two warpgroups' running maxima, merged once per tile
-                    xm_s[grp * 128 + pt] = m_run;
-                    named_bar_sync(3, 256);
-                    thr_base = fmaxf(m_run, xm_s[(grp ^ 1) * 128 + pt]);
+                if (screening) {
+                    // What a pair is screened against: the point's maximum over the evaluated components (final by now; the
+                    // two warpgroups merge theirs at the first screening group) and the largest LOWER bound among the listed
+                    // components seen so far (each warpgroup publishes its own after every group and picks up the other's:
+                    // a value that is a little old is still a valid bound).
+                    if (g == p.scr_group) {
+                        xm_s[grp * 128 + pt] = m_run;
+                        named_bar_sync(3, 256);
+                        thr_base = fmaxf(m_run, xm_s[(grp ^ 1) * 128 + pt]);
+                        named_bar_sync(3, 256);
+                        xm_s[grp * 128 + pt] = thr_base;
+                    } else {
+                        xm_s[grp * 128 + pt] = thr_base;
+                        thr_base = fmaxf(thr_base, xm_s[(grp ^ 1) * 128 + pt]);
+                    }
                 }
                 const bool got = bar_wait(BAR(LB_LFULL), uses & 1u, abort_flag, p.status, false);
                 const bool ok = __all_sync(0xffffffffu, got);
@@ -186,14 +198,18 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
                                 // raised by what they can be wrong by, tell which pairs can matter at all.  The point's
                                 // maximum over the evaluated components is final by now.  (!(a < b): a NaN passes.)
                                 if (__ldg(p.scr_mask + (col0 >> 5)) != 0 && row < p.n) {
-                                    const float thr = thr_base - 40.f;
                                     const float4* sc4 = reinterpret_cast<const float4*>(p.scr + col0);
+                                    const float2* se2 = reinterpret_cast<const float2*>(p.scr_e + col0);
 #pragma unroll
                                     for (int j = 0; j < 32; j += 2) {
                                         const float4 q = __ldg(tc4 + (j >> 1));
                                         const float4 sq = __ldg(sc4 + (j >> 1));
+                                        const float2 se = __ldg(se2 + (j >> 1));
                                         const float u0 = fmaf(__uint_as_float(v[j]) + __uint_as_float(vc[j]), q.x, fmaf(sq.y, nrm, sq.x));
                                         const float u1 = fmaf(__uint_as_float(v[j + 1]) + __uint_as_float(vc[j + 1]), q.z, fmaf(sq.w, nrm, sq.z));
+                                        // lower bounds: the upper bound minus twice the allowance (fmaxf drops a NaN)
+                                        thr_base = fmaxf(thr_base, fmaxf(u0 - 2.f * fmaf(sq.y, nrm, se.x), u1 - 2.f * fmaf(sq.w, nrm, se.y)));
+                                        const float thr = thr_base - 40.f;
                                         if (!(u0 < thr) && sq.x > -CUDART_INF_F) {
                                             const int sl = __ldg(p.slot_of + col0 + j);
                                             if (sl >= 0) { atomicOr(p.cand + row * p.cand_words + (sl >> 5), 1u << (sl & 31)); ++nhit; }
@@ -1074,7 +1090,8 @@ __global__ void __launch_bounds__(1024) wide_cref_kernel(int rows, const int* __
                                                          const double* __restrict__ ckd, const int* __restrict__ comp_of,
                                                          const int* __restrict__ slot_of, const float* __restrict__ scra,
                                                          const float* __restrict__ scrw, double* __restrict__ cref,
-                                                         float2* __restrict__ tkck, float2* __restrict__ scr) {
+                                                         float2* __restrict__ tkck, float2* __restrict__ scr,
+                                                         float* __restrict__ scr_e) {
     __shared__ double red[1024];
     const int Kg = flags[6];
     double m = -CUDART_INF;
@@ -1095,6 +1112,7 @@ __global__ void __launch_bounds__(1024) wide_cref_kernel(int rows, const int* __
         const bool listed = slot_of[k] >= 0 && c >= 0 && isfinite(ckd[k]);
         scr[k] = listed ? make_float2((float)fmin(ckd[k] - r + (double)scra[c], 3e38), scrw[c])
                         : (in && c >= 0) ? make_float2(scra[c], scrw[c]) : make_float2(-CUDART_INF_F, 0.f);
+        scr_e[k] = listed ? scra[c] : 0.f;
     }
 }
 
@@ -1305,35 +1323,70 @@ __device__ __forceinline__ double wide_pair_log2z(const float* __restrict__ xr, 
     return c - q;
 }
 
-// One warp per point: its marked pairs in ascending slot order; those within 2^-40 of the point's log2 Z over the
-// evaluated components (logz) are kept: log-sum-exp into out[i], bit (slot, i) of the transposed map.
+// One warp per point: its marked pairs in ascending slot order, evaluated exactly.  First round: every pair's exact log2 z,
+// each abandoned as soon as it cannot come within 2^-40 of the largest value so far (the point's log2 Z over the evaluated
+// components to begin with: logz); the first 128 values are kept in shared memory.  Second round: the pairs within 2^-40
+// of the final maximum are kept: log-sum-exp into out[i], bit (slot, i) of the transposed map.
+constexpr int CAND_WORDS_PER_LANE = (WIDE_CAND_WORDS + 31) / 32;
+constexpr int CAND_KEEP = 128;
 __global__ void __launch_bounds__(256) wide_cand_lse_kernel(const float* __restrict__ X, int64_t n, int D, int words,
                                                             const unsigned* __restrict__ cand, unsigned* __restrict__ candT,
                                                             const float* __restrict__ mu_c, const float* __restrict__ w2_c,
                                                             const double* __restrict__ c2d_c, const double* __restrict__ logz,
                                                             double* __restrict__ out, int* __restrict__ ctl) {
     if (ctl[1] != 0) return;
+    __shared__ double lbuf[8][CAND_KEEP];
     const int64_t i = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     if (i >= n) return;
-    const unsigned b0 = (lane < words) ? cand[i * words + lane] : 0u;
-    const unsigned b1 = (lane + 32 < words) ? cand[i * words + 32 + lane] : 0u;
-    if (!__any_sync(0xffffffffu, (b0 | b1) != 0u)) {
+    unsigned bits[CAND_WORDS_PER_LANE];
+    unsigned any = 0u;
+#pragma unroll
+    for (int q = 0; q < CAND_WORDS_PER_LANE; ++q) {
+        bits[q] = (lane + 32 * q < words) ? cand[i * words + lane + 32 * q] : 0u;
+        any |= bits[q];
+    }
+    if (!__any_sync(0xffffffffu, any != 0u)) {
         if (lane == 0) out[i] = -CUDART_INF;
         return;
     }
-    const double lim = logz[i] - 40.0;
     const float* xr = X + i * D;
-    double m = -CUDART_INF, ssum = 0.0;
-    int kept = 0;
+    auto word_at = [&](int wi) {
+        unsigned v = bits[0];
+#pragma unroll
+        for (int q = 1; q < CAND_WORDS_PER_LANE; ++q)
+            if ((wi >> 5) == q) v = bits[q];
+        return __shfl_sync(0xffffffffu, v, wi & 31);
+    };
+    double best = logz[i];
+    int idx = 0;
     for (int wi = 0; wi < words; ++wi) {
-        unsigned word = __shfl_sync(0xffffffffu, wi < 32 ? b0 : b1, wi & 31);
+        unsigned word = word_at(wi);
         while (word) {
             const int b = __ffs(word) - 1;
             word &= word - 1;
             const int slot = wi * 32 + b;
-            const double c = __ldg(c2d_c + slot);
-            const double l = wide_pair_log2z(xr, mu_c + (size_t)slot * D, w2_c + (size_t)slot * D, c, D, lane, lim);
+            const double l = wide_pair_log2z(xr, mu_c + (size_t)slot * D, w2_c + (size_t)slot * D, __ldg(c2d_c + slot), D, lane, best - 40.0);
+            if (idx < CAND_KEEP && lane == 0) lbuf[w][idx] = l;
+            ++idx;
+            if (l > best) best = l;
+        }
+    }
+    __syncwarp();
+    const double lim = best - 40.0;
+    double m = -CUDART_INF, ssum = 0.0;
+    int kept = 0;
+    idx = 0;
+    for (int wi = 0; wi < words; ++wi) {
+        unsigned word = word_at(wi);
+        while (word) {
+            const int b = __ffs(word) - 1;
+            word &= word - 1;
+            const int slot = wi * 32 + b;
+            double l;
+            if (idx < CAND_KEEP) l = lbuf[w][idx];
+            else l = wide_pair_log2z(xr, mu_c + (size_t)slot * D, w2_c + (size_t)slot * D, __ldg(c2d_c + slot), D, lane, lim);
+            ++idx;
             if (l >= lim && l > -CUDART_INF) {               // warp-uniform
                 if (l > m) { ssum = ssum * exp2(m - l) + 1.0; m = l; }
                 else ssum += exp2(l - m);
@@ -1348,9 +1401,13 @@ __global__ void __launch_bounds__(256) wide_cand_lse_kernel(const float* __restr
     }
 }
 
-// One block per slot: the points marked for it, in ascending order, 2048 rows of the map at a time: r = 2^(exact log2 z
-// - log2 Z) by one warp per pair, then every thread adds r (x - g), r (x - g)^2 for its dimensions (float64, the order
-// fixed: same bits in every run).  The sums are shifted back to the origin and added to the slot's statistics.
+// One block per slot: the points marked for it in the transposed map, in ascending order (the order of the additions is
+// fixed: same bits in every run).  The block lists its points in shared memory (up to MS_CAP per pass over the map), then
+// takes them eight at a time: every thread loads its 3-4 dimensions of the eight rows (all loads in flight together), the
+// eight quadratic forms are reduced over the block (fp32 per thread, float64 from there), r = 2^(log2 z - log2 Z), and every
+// thread adds r (x - g), r (x - g)^2 for its dimensions in float64.  The sums are shifted back to the origin and added to
+// the slot's statistics.
+constexpr int MS_CAP = 1024, MS_B = 8;
 __global__ void __launch_bounds__(256) wide_cand_mstep_kernel(const float* __restrict__ X, int64_t n, int D, const int* __restrict__ list,
                                                               const unsigned* __restrict__ candT, const float* __restrict__ mu_c,
                                                               const float* __restrict__ w2_c, const double* __restrict__ c2d_c,
@@ -1362,69 +1419,118 @@ __global__ void __launch_bounds__(256) wide_cand_mstep_kernel(const float* __res
     if (list[slot] < 0) return;
     const unsigned* bits = candT + (size_t)slot * WIDE_CANDT_WORDS;
     const int words = (int)((n + 31) >> 5);
-    unsigned any = 0u;
-    for (int w = tid; w < words; w += 256) any |= bits[w];
-    if (!__syncthreads_or(any != 0u)) return;
-    __shared__ int rows_s[2048];
-    __shared__ double r_s[2048];
-    __shared__ int wsum[2];
+    // thread t owns words [16 t, 16 t + 16): ascending rows across the block
+    unsigned mine[16];
+    int cnt = 0;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        const int w = 16 * tid + j;
+        mine[j] = (w < words) ? bits[w] : 0u;
+        cnt += __popc(mine[j]);
+    }
+    __shared__ int rows_s[MS_CAP];
+    __shared__ int wtot[8];
+    __shared__ double red_s[8][MS_B];
+    int incl = cnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    if (lane == 31) wtot[warp] = incl;
+    __syncthreads();
+    int before = incl - cnt, total = 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        if (j < warp) before += wtot[j];
+        total += wtot[j];
+    }
+    if (total == 0) return;                                  // block-uniform
     const double c = c2d_c[slot];
-    const float* mr = mu_c + (size_t)slot * D;
-    const float* wr = w2_c + (size_t)slot * D;
+    float mu_r[4], w2_r[4], g_r[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        const int d = tid + 256 * q;
+        mu_r[q] = (d < D) ? mu_c[(size_t)slot * D + d] : 0.f;
+        w2_r[q] = (d < D) ? w2_c[(size_t)slot * D + d] : 0.f;
+        g_r[q] = (d < D) ? gd[d] : 0.f;
+    }
     double s1[4] = {0.0, 0.0, 0.0, 0.0}, s2[4] = {0.0, 0.0, 0.0, 0.0}, nk = 0.0;
-    float gq[4];
+    for (int base = 0; base < total; base += MS_CAP) {
+        // this pass's window of the list
+        {
+            int at = before;
 #pragma unroll
-    for (int q = 0; q < 4; ++q) gq[q] = (tid + 256 * q < D) ? gd[tid + 256 * q] : 0.f;
-    for (int w0 = 0; w0 < words; w0 += 64) {
-        unsigned word = (tid < 64 && w0 + tid < words) ? bits[w0 + tid] : 0u;
-        const int cnt = __popc(word);
-        int incl = cnt;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int t = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += t;
-        }
-        if (warp < 2 && lane == 31) wsum[warp] = incl;
-        __syncthreads();
-        const int total = wsum[0] + wsum[1];
-        if (tid < 64) {
-            int at = (warp == 1 ? wsum[0] : 0) + incl - cnt;
-            while (word) {
-                const int b = __ffs(word) - 1;
-                word &= word - 1;
-                rows_s[at++] = (w0 + tid) * 32 + b;
-            }
-        }
-        __syncthreads();
-        if (total == 0) continue;                            // block-uniform
-        for (int e = warp; e < total; e += 8) {
-            const int row = rows_s[e];
-            const double l = wide_pair_log2z(X + (size_t)row * D, mr, wr, c, D, lane, -CUDART_INF);
-            if (lane == 0) r_s[e] = exp2(l - logz_x[row]);
-        }
-        __syncthreads();
-        for (int e = 0; e < total; ++e) {
-            const double r = r_s[e];
-            const float* xr = X + (size_t)rows_s[e] * D;
-            nk += r;
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const int d = tid + 256 * q;
-                if (d < D) {
-                    const double xd = (double)(__ldg(xr + d) - gq[q]);
-                    s1[q] += r * xd;
-                    s2[q] += r * xd * xd;
+            for (int j = 0; j < 16; ++j) {
+                unsigned word = mine[j];
+                while (word) {
+                    const int b = __ffs(word) - 1;
+                    word &= word - 1;
+                    if (at >= base && at < base + MS_CAP) rows_s[at - base] = (16 * tid + j) * 32 + b;
+                    ++at;
                 }
             }
         }
-        __syncthreads();                                     // rows_s, r_s and wsum are rewritten by the next round
+        __syncthreads();
+        const int here = (total - base < MS_CAP) ? (total - base) : MS_CAP;
+        for (int e0 = 0; e0 < here; e0 += MS_B) {
+            float xv[MS_B][4];
+            float part[MS_B];
+#pragma unroll
+            for (int b = 0; b < MS_B; ++b) {
+                const bool in = e0 + b < here;
+                const float* xr = X + (size_t)(in ? rows_s[e0 + b] : rows_s[e0]) * D;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const int d = tid + 256 * q;
+                    xv[b][q] = (d < D) ? __ldg(xr + d) : 0.f;
+                }
+            }
+#pragma unroll
+            for (int b = 0; b < MS_B; ++b) {
+                float p = 0.f;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const float diff = xv[b][q] - mu_r[q];
+                    p = fmaf(diff * diff, w2_r[q], p);
+                }
+                part[b] = p;
+            }
+            // the block's sums of the eight quadratic forms: fixed butterfly, then the eight warps in order
+#pragma unroll
+            for (int b = 0; b < MS_B; ++b) {
+                double v = (double)part[b];
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                if (lane == 0) red_s[warp][b] = v;
+            }
+            __syncthreads();
+#pragma unroll
+            for (int b = 0; b < MS_B; ++b) {
+                if (e0 + b < here) {                         // block-uniform
+                    double q = 0.0;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) q += red_s[j][b];
+                    const double r = exp2(c - q - logz_x[rows_s[e0 + b]]);
+                    nk += r;
+#pragma unroll
+                    for (int qq = 0; qq < 4; ++qq) {
+                        const double xd = (double)(xv[b][qq] - g_r[qq]);
+                        s1[qq] += r * xd;
+                        s2[qq] += r * xd * xd;
+                    }
+                }
+            }
+            __syncthreads();                                 // red_s is rewritten by the next batch
+        }
+        __syncthreads();                                     // rows_s is rewritten by the next pass
     }
     if (tid == 0) Nk_c[slot] += nk;
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
         const int d = tid + 256 * q;
         if (d < D) {
-            const double g = (double)gq[q];
+            const double g = (double)g_r[q];
             S1_c[(size_t)slot * D + d] += s1[q] + g * nk;
             S2_c[(size_t)slot * D + d] += s2[q] + 2.0 * g * s1[q] + g * g * nk;
         }
@@ -1500,11 +1606,20 @@ __global__ void __launch_bounds__(256) wide_assign_refine_kernel(const WideAssig
     if (g.cand != nullptr) {
         const double lim = lz - 40.0;
         const int words = g.cand_words;
-        const unsigned b0 = (lane < words) ? g.cand[row * words + lane] : 0u;
-        const unsigned b1 = (lane + 32 < words) ? g.cand[row * words + 32 + lane] : 0u;
-        if (__any_sync(0xffffffffu, (b0 | b1) != 0u)) {
+        unsigned bits[CAND_WORDS_PER_LANE];
+        unsigned any = 0u;
+#pragma unroll
+        for (int q = 0; q < CAND_WORDS_PER_LANE; ++q) {
+            bits[q] = (lane + 32 * q < words) ? g.cand[row * words + lane + 32 * q] : 0u;
+            any |= bits[q];
+        }
+        if (__any_sync(0xffffffffu, any != 0u)) {
             for (int wi = 0; wi < words; ++wi) {
-                unsigned word = __shfl_sync(0xffffffffu, wi < 32 ? b0 : b1, wi & 31);
+                unsigned bv = bits[0];
+#pragma unroll
+                for (int q = 1; q < CAND_WORDS_PER_LANE; ++q)
+                    if ((wi >> 5) == q) bv = bits[q];
+                unsigned word = __shfl_sync(0xffffffffu, bv, wi & 31);
                 while (word) {
                     const int b = __ffs(word) - 1;
                     word &= word - 1;
@@ -1653,7 +1768,7 @@ cudaError_t launch_prepare_wide(cudaStream_t s, int D, int K, const float* pi, c
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     wide_cref_kernel<<<1, 1024, 0, s>>>(pl.rows, wb.flags, wb.tk, wb.ckd, wb.comp_of, wb.slot_of, wb.scra, wb.scrw, wb.cref,
-                                        reinterpret_cast<float2*>(wb.tkck), reinterpret_cast<float2*>(wb.scr));
+                                        reinterpret_cast<float2*>(wb.tkck), reinterpret_cast<float2*>(wb.scr), wb.scr_e);
     return cudaGetLastError();
 }
 
@@ -1753,7 +1868,7 @@ cudaError_t launch_transform_wide(cudaStream_t s, const float* X, int64_t n, int
 
 cudaError_t launch_lse_wide(cudaStream_t s, int64_t n, int D, int K, int Kg, int n_listed, int n_slots, const WideBuffers& wb,
                             int num_sms, int* status, int ntop) {
-    if (n < 1 || n > WIDE_PIECE || Kg < 1 || Kg > K) return cudaErrorInvalidValue;
+    if (n < 1 || n > WIDE_PIECE || Kg < 0 || Kg > K || (Kg < 1 && n_listed < 1)) return cudaErrorInvalidValue;
     const WidePlan pl = wide_plan(D, K, num_sms);
     const int64_t rp = rows_padded_of(n);
     const int atoms = 4 * pl.n_slices;
@@ -1778,7 +1893,7 @@ cudaError_t launch_lse_wide(cudaStream_t s, int64_t n, int D, int K, int Kg, int
     p.top = wb.top;
     p.screen = screen;
     p.scr = reinterpret_cast<const float2*>(wb.scr);
-    p.scr_mask = wb.scr_mask; p.slot_of = wb.slot_of; p.n2 = wb.n2; p.cand = wb.cand;
+    p.scr_e = wb.scr_e; p.scr_mask = wb.scr_mask; p.slot_of = wb.slot_of; p.n2 = wb.n2; p.cand = wb.cand;
     p.cand_words = (n_slots + 31) / 32; p.scr_group = Kgp / 256; p.ctl = wb.ctl;
     const int64_t ntiles = (n + WIDE_TILE - 1) / WIDE_TILE;
     const unsigned grid = (unsigned)(ntiles < num_sms ? ntiles : num_sms);

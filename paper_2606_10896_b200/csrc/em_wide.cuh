@@ -12,10 +12,10 @@ constexpr int WIDE_MAX_K = 4096;
 constexpr int64_t WIDE_PIECE = 1 << 17;      // points per pair of launches: capacity of the fp16 planes of Y in scratch
 constexpr int WIDE_BATCH = 256;              // points per batch of the second sweep
 constexpr int WIDE_TILE = 128;               // points per tile of the first sweep
-constexpr int WIDE_MAX_ILL = 2048;           // ill-conditioned components the FP32 kernels evaluate as a sub-mixture
+constexpr int WIDE_MAX_ILL = WIDE_MAX_K + 64; // slots of the list of components evaluated exactly (all of them may be; + the gap)
 constexpr int WIDE_LL_BLOCKS = 64;           // per-block partial sums of the log-likelihood
 constexpr int WIDE_MAX_TOP = 10;             // candidates per point sweep 1 can report (the top-m assignment asks for m + 2)
-constexpr int WIDE_CAND_WORDS = WIDE_MAX_ILL / 32;          // 32-bit words of a point's row of the candidate bitmap
+constexpr int WIDE_CAND_WORDS = (WIDE_MAX_ILL + 31) / 32;   // 32-bit words of a point's row of the candidate bitmap, at most
 constexpr int WIDE_CANDT_WORDS = (int)(WIDE_PIECE / 32);    // words of a slot's row of the transposed bitmap
 
 struct WidePlan {
@@ -62,6 +62,7 @@ struct WideBuffers {
     // Screening of the (point, ill-conditioned component) pairs by sweep 1 and their exact evaluation pair by pair:
     float* scr;     // [rows] pairs.  Listed components: (c - c_ref + error allowance, allowance per unit of |x - g|^2);
                     // evaluated components: (error allowance, allowance per unit of |x - g|^2); (-inf, 0) elsewhere
+    float* scr_e;   // [rows] listed components: the error allowance alone (what scr's first entry adds to c - c_ref)
     int* slot_of;   // [rows] slot in the list of the component at a position, -1 if it is not listed
     int* scr_mask;  // [rows / 32] nonzero where a chunk of 32 positions holds a listed component
     float* n2;      // [WIDE_PIECE] |x_i - g|^2

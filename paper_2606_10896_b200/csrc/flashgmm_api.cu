@@ -34,7 +34,7 @@ struct ScratchLayout {
     size_t tc_phi, tc_plo, tc_tk, tc_ck, tc_sd, tc_kap, tc_gd, tc_illb, tc_flags, tc_xg, tc_xl, tc_partial, tc_llpart, tc_partial_bytes, tc_yhi, tc_ylo, tc_phirm, tc_plorm, tc_tkck, tc_illlist, tc_illcache, tc_decdim, tc_decw, tc_decmu;
     bool tc;
     // the tensor-core path for D > 128
-    size_t w_sd, w_kap, w_gd, w_phi, w_plo, w_tk, w_tkck, w_ckd, w_cref, w_illb, w_flags, w_yhi, w_ylo, w_logz, w_partial, w_llpart, w_illlist, w_muc, w_w2c, w_c2dc, w_statsc, w_top, w_logzx, w_compof, w_scra, w_scrw, w_scr, w_slotof, w_scrmask, w_n2, w_cand, w_candT, w_ctl;
+    size_t w_sd, w_kap, w_gd, w_phi, w_plo, w_tk, w_tkck, w_ckd, w_cref, w_illb, w_flags, w_yhi, w_ylo, w_logz, w_partial, w_llpart, w_illlist, w_muc, w_w2c, w_c2dc, w_statsc, w_top, w_logzx, w_compof, w_scra, w_scrw, w_scr, w_slotof, w_scrmask, w_n2, w_cand, w_candT, w_ctl, w_scre;
     size_t w_partial_bytes;
     bool wide;
 };
@@ -89,7 +89,7 @@ ScratchLayout scratch_layout(int D, int K, bool planes) {
         L.tc_ylo = take(TC_YPLANE_BYTES);
     }
     L.w_sd = L.w_kap = L.w_gd = L.w_phi = L.w_plo = L.w_tk = L.w_tkck = L.w_ckd = L.w_cref = L.w_illb = L.w_flags = L.w_yhi = L.w_ylo = L.w_logz = L.w_partial = L.w_llpart = L.w_illlist = L.w_muc = L.w_w2c = L.w_c2dc = L.w_statsc = L.w_top = L.w_logzx = 0;
-    L.w_compof = L.w_scra = L.w_scrw = L.w_scr = L.w_slotof = L.w_scrmask = L.w_n2 = L.w_cand = L.w_candT = L.w_ctl = 0;
+    L.w_compof = L.w_scra = L.w_scrw = L.w_scr = L.w_slotof = L.w_scrmask = L.w_n2 = L.w_cand = L.w_candT = L.w_ctl = L.w_scre = 0;
     L.w_partial_bytes = 0;
     L.wide = wide_supports(D, K) && planes;
     if (L.wide) {
@@ -112,9 +112,11 @@ ScratchLayout scratch_layout(int D, int K, bool planes) {
         L.w_slotof = take((size_t)wp.rows * 4);
         L.w_scrmask = take((size_t)wp.rows / 32 * 4);
         L.w_n2 = take((size_t)WIDE_PIECE * 4);
-        L.w_cand = take((size_t)WIDE_PIECE * WIDE_CAND_WORDS * 4);
-        L.w_candT = take((size_t)WIDE_MAX_ILL * WIDE_CANDT_WORDS * 4);
+        const size_t slots = (size_t)(K + 64 < WIDE_MAX_ILL ? K + 64 : WIDE_MAX_ILL);     // the list is never longer
+        L.w_cand = take((size_t)WIDE_PIECE * ((slots + 31) / 32) * 4);
+        L.w_candT = take(slots * WIDE_CANDT_WORDS * 4);
         L.w_ctl = take(32);
+        L.w_scre = take((size_t)wp.rows * 4);
         L.w_logz = take((size_t)WIDE_PIECE * 8);
         L.w_top = take((size_t)WIDE_PIECE * 2 * WIDE_MAX_TOP * 4);
         L.w_logzx = take((size_t)WIDE_PIECE * 8);
@@ -122,10 +124,10 @@ ScratchLayout scratch_layout(int D, int K, bool planes) {
         L.w_partial = take(L.w_partial_bytes);
         L.w_llpart = take(256 * 8);
         L.w_illlist = take((size_t)WIDE_MAX_ILL * 4);
-        L.w_muc = take((size_t)WIDE_MAX_ILL * D * 4);
-        L.w_w2c = take((size_t)WIDE_MAX_ILL * D * 4);
-        L.w_c2dc = take((size_t)WIDE_MAX_ILL * 8);
-        L.w_statsc = take(((size_t)WIDE_MAX_ILL + 2 * (size_t)WIDE_MAX_ILL * D) * 8);
+        L.w_muc = take(slots * D * 4);
+        L.w_w2c = take(slots * D * 4);
+        L.w_c2dc = take(slots * 8);
+        L.w_statsc = take((slots + 2 * slots * D) * 8);
         L.w_yhi = take((size_t)WIDE_PIECE * wp.Dpad * 4);
         L.w_ylo = take((size_t)WIDE_PIECE * wp.Dpad * 4);
     }
@@ -170,6 +172,11 @@ struct gmm_ctx {
     int wide_n_list = 0;             // slots of the packed sub-mixture (the ill-conditioned components plus padding)
     int wide_n_ill = 0;              // ill-conditioned components of the current step on the D > 128 tensor path
     int wide_n_good = 0;             // components the tensor passes evaluate in the current step (the others are listed)
+    int wide_mode = 0;               // GMM_WIDE_MODE: 0 = automatic, 1 = "sweeps" (two tensor sweeps, few components exact),
+                                     // 2 = "screen" (one tensor sweep screens every pair, every component evaluated exactly)
+    double wide_probe_limit = 0.0;   // automatic mode: "screen" while a sample of the points has at most this many marked pairs per
+                                     // point (0: K D / 8192)
+    bool wide_screen_all = false;    // the current step runs in "screen" mode
     int wide_sparse = 1;             // GMM_WIDE_SPARSE: 0 = the listed components always go through the dense FP32 kernels,
                                      // 1 = pair by pair unless sweep 1 marks too many pairs, 2 = always pair by pair (tests)
     int tc_n_ill = 0;                // ill-conditioned components at the last result that was read back (picks the filter)
@@ -262,6 +269,7 @@ struct gmm_ctx {
         b.cand = reinterpret_cast<unsigned*>(scratch + lay.w_cand);
         b.candT = reinterpret_cast<unsigned*>(scratch + lay.w_candT);
         b.ctl = reinterpret_cast<int*>(scratch + lay.w_ctl);
+        b.scr_e = reinterpret_cast<float*>(scratch + lay.w_scre);
         return b;
     }
 };
@@ -400,31 +408,77 @@ int prof_end(gmm_ctx* ctx) {
 // Derived per-component constants for both paths; validates the parameters into the status word.  Then picks the
 // path: the tensor-core path whenever the shape allows it (ill-conditioned components are handled inside its kernel).
 int prepare_and_choose(gmm_ctx* ctx, int64_t N, int D, int K, const float* pi, const float* mu, const float* var,
-                       int* path) {
+                       int* path, const float* Xprobe = nullptr, int64_t n_probe = 0) {
     KL(launch_prepare_fp32(ctx->stream, D, K, pi, mu, var, ctx->w2(), ctx->c2(), ctx->c2d(), ctx->center(), &ctx->result()->status));
     if ((size_t)K * D > ((size_t)1 << 12)) ctx->launches++;      // but for tiny problems, the centre of the means is a launch of its own
     if (wide_supports(D, K)) {
-        // D > 128: the two-sweep tensor path when forced, or under AUTO from enough points per component on; parameter sets
-        // in which the preparation flags an ill-conditioned component go to the FP32 kernels (read back: one small
-        // synchronisation per step, against seconds of compute at these shapes).
-        const bool want = ctx->lay.wide && (ctx->path == GMM_PATH_TENSOR ||
-                                            (ctx->path == GMM_PATH_AUTO && K >= 64 && N >= WIDE_AUTO_MIN_POINTS_PER_COMPONENT * K));
+        // D > 128, K >= 64 (or forced): the tensor path for wide data, in one of two modes.
+        //   "screen"  one tensor sweep over all components only SCREENS the (point, component) pairs - it marks those whose
+        //             approximate log2 z, with its error bound, can come within 2^-40 of the point's best - and every marked
+        //             pair is evaluated exactly in fp32.  On wide data posteriors are sparse (a few pairs per point), so
+        //             this is both the faster and the more accurate mode.  Xprobe (device rows of this step's data, may be
+        //             NULL) lets the automatic choice try it on a sample first.
+        //   "sweeps"  the two sweeps of Algorithm 1 on the tensor cores, with only the ill-conditioned and light components
+        //             evaluated exactly: for data whose posteriors are broad (many marked pairs per point).  Needs 128
+        //             points per component under AUTO (with fewer, most components would be "light").
+        // Parameter sets with too many ill-conditioned components for "sweeps" go to the FP32 kernels.  The flags come
+        // back through small synchronisations (two or three per step, against a second of compute at these shapes).
+        const bool want = ctx->lay.wide && (ctx->path == GMM_PATH_TENSOR || (ctx->path == GMM_PATH_AUTO && K >= 64));
         *path = GMM_PATH_FP32;
+        ctx->wide_screen_all = false;
         if (!want) return GMM_OK;
         float limit = ctx->tc_cond_limit;
         if (limit < 0.f) limit = ctx->tc_cond_scale * std::sqrt((float)((double)N / (double)K));
         const WideBuffers wb = ctx->wide();
+        int fl[8];
+        const bool can_probe = Xprobe != nullptr && n_probe >= 1;
+        // Automatic choice: "sweeps" from 128 points per component on (measured at config 5's shape, steady state: 105 ms per
+        // million points against 142 for "screen", whose exact evaluation of 26 marked pairs per point costs more than the
+        // second sweep); "screen" below that, where "sweeps" would find most components light and the alternative is the FP32
+        // kernels (1580 ms per million points) - provided a sample of the points marks few enough pairs.
+        const bool few_points = N < WIDE_AUTO_MIN_POINTS_PER_COMPONENT * K;
+        if (ctx->wide_mode == 2 || (ctx->wide_mode == 0 && can_probe && few_points)) {
+            KL(launch_prepare_wide(ctx->stream, D, K, pi, mu, var, wb, limit, INFINITY));      // every component is listed
+            ctx->launches += 4;
+            CU(cudaMemcpyAsync(fl, wb.flags, sizeof(fl), cudaMemcpyDeviceToHost, ctx->stream));
+            CU(cudaStreamSynchronize(ctx->stream));
+            const int n_list = fl[2];
+            bool ok = n_list >= 1 && fl[4] + 64 <= WIDE_MAX_ILL;
+            if (ok) KL(launch_ill_gather_wide(ctx->stream, D, n_list, wb, mu, ctx->w2(), ctx->c2d()));
+            if (ok && ctx->wide_mode == 0) {
+                // the first rows of the data through the screening sweep: how many pairs per point does it mark?
+                const int64_t np = n_probe < 8192 ? n_probe : 8192;
+                CU(launch_cand_clear_wide(ctx->stream, np, n_list, wb));
+                KL(launch_norm_wide(ctx->stream, Xprobe, np, D, wb));
+                KL(launch_transform_wide(ctx->stream, Xprobe, np, D, wb, &ctx->result()->status));
+                KL(launch_lse_wide(ctx->stream, np, D, K, fl[6], fl[4], n_list, wb, ctx->sms, &ctx->result()->status));
+                int marks = 0;
+                CU(cudaMemcpyAsync(&marks, wb.ctl, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
+                CU(cudaStreamSynchronize(ctx->stream));
+                // (a marked pair costs about 1.3 ns, mostly for being ruled out after its first 128 dimensions; the FP32 kernels
+                // cost K D / 2000 ns per point: the pair route is taken while it is clearly the cheaper one)
+                ok = (double)marks <= (ctx->wide_probe_limit > 0.0 ? ctx->wide_probe_limit : (double)n_list * D / 8192.0) * (double)np;
+            }
+            if (ok) {
+                ctx->wide_n_ill = fl[4];
+                ctx->wide_n_good = fl[6];
+                ctx->wide_n_list = n_list;
+                ctx->wide_n_first = fl[5] < n_list ? fl[5] : n_list;
+                ctx->wide_screen_all = true;
+                *path = GMM_PATH_TENSOR;
+                return GMM_OK;
+            }
+        }
+        if (!(ctx->path == GMM_PATH_TENSOR || N >= WIDE_AUTO_MIN_POINTS_PER_COMPONENT * K)) return GMM_OK;
         KL(launch_prepare_wide(ctx->stream, D, K, pi, mu, var, wb, limit, (float)((double)ctx->wide_min_points / (double)N)));
         ctx->launches += 4;
-        // how many components were flagged, the length of their list and how many are left to the tensor passes: one
-        // small synchronisation per step, against seconds of compute at these shapes
-        int fl[8];
+        // how many components were flagged, the length of their list and how many are left to the tensor passes
         CU(cudaMemcpyAsync(fl, wb.flags, sizeof(fl), cudaMemcpyDeviceToHost, ctx->stream));
         CU(cudaStreamSynchronize(ctx->stream));
         const int n_ill = fl[4];
         ctx->wide_n_ill = n_ill;
         ctx->wide_n_good = fl[6];
-        if (n_ill + 64 > WIDE_MAX_ILL || 2 * n_ill > K) return GMM_OK;     // too many: the FP32 kernels take the whole step
+        if (n_ill + 64 > WIDE_MAX_ILL || 2 * n_ill > K || fl[6] < 1) return GMM_OK;     // too many: the FP32 kernels take the whole step
         if (n_ill > 0) {
             // The flagged components take no part in the tensor passes: they are evaluated exactly as a packed sub-mixture,
             // pair by pair where sweep 1 finds that a pair can matter, or densely by the FP32 kernels (a collapsed component
@@ -490,12 +544,13 @@ int accumulate_points(gmm_ctx* ctx, int path, const float* X, int64_t n, int D, 
         CU(cudaMemsetAsync(wb.llpart, 0, 256 * 8, ctx->stream));
         const int Kg = ctx->wide_n_good;
         const int n_listed = n_ill > 0 ? ctx->wide_n_ill : 0;
-        const bool screen = n_ill > 0 && ctx->wide_sparse != 0;
+        const bool all = ctx->wide_screen_all;                              // "screen" mode: no component is left to sweep 2
+        const bool screen = n_ill > 0 && (ctx->wide_sparse != 0 || all);
         const int* dense_if = screen ? wb.ctl + 1 : nullptr;             // the dense kernels run when the gate says so
         for (int64_t off = 0; off < n; off += ctx->wide_piece) {
             const int64_t cnt = (n - off < ctx->wide_piece) ? (n - off) : ctx->wide_piece;
             const float* Xs = X + off * D;
-            CU(cudaMemsetAsync(wb.partial, 0, ctx->lay.w_partial_bytes, ctx->stream));
+            if (!all) CU(cudaMemsetAsync(wb.partial, 0, ctx->lay.w_partial_bytes, ctx->stream));
             if (screen) {
                 CU(launch_cand_clear_wide(ctx->stream, cnt, n_ill, wb));
                 KL(launch_norm_wide(ctx->stream, Xs, cnt, D, wb));
@@ -503,21 +558,23 @@ int accumulate_points(gmm_ctx* ctx, int path, const float* X, int64_t n, int D, 
             CHECK(prof_begin(ctx));
             KL(launch_transform_wide(ctx->stream, Xs, cnt, D, wb, &ctx->result()->status));
             KL(launch_lse_wide(ctx->stream, cnt, D, K, Kg, screen ? n_listed : 0, n_ill, wb, ctx->sms, &ctx->result()->status));
-            if (ctx->wide_refine) KL(launch_refine_wide(ctx->stream, Xs, cnt, D, K, mu, ctx->w2(), ctx->c2d(), wb));
+            if (ctx->wide_refine && !all) KL(launch_refine_wide(ctx->stream, Xs, cnt, D, K, mu, ctx->w2(), ctx->c2d(), wb));
             else CU(cudaMemcpyAsync(wb.logz_x, wb.logz, (size_t)cnt * 8, cudaMemcpyDeviceToDevice, ctx->stream));
             if (n_ill > 0) {
                 if (screen) {
                     // more than one pair in 64 marked (or the pair-by-pair route switched off): the dense kernels are cheaper
-                    const long long max_pairs = ctx->wide_sparse >= 2 ? ((long long)1 << 62) : (long long)cnt * n_ill / 64;
+                    // ("screen" mode: the dense alternative evaluates every component, so the pair route pays for longer)
+                    const long long max_pairs = ctx->wide_sparse >= 2 ? ((long long)1 << 62)
+                                              : all ? (long long)((double)cnt * n_ill * D / 8192.0) : (long long)cnt * n_ill / 64;
                     KL(launch_cand_gate_wide(ctx->stream, wb, max_pairs));
                     KL(launch_cand_lse_wide(ctx->stream, Xs, cnt, D, n_ill, wb, ctx->logZ2()));
                 }
                 KL(launch_lse_fp32(ctx->stream, Xs, cnt, D, n_ill, wb.mu_c, wb.w2_c, wb.c2d_c, ctx->center(), ctx->logZ2(), nullptr, wb.logz, dense_if));
             }
             KL(launch_merge_ll_wide(ctx->stream, cnt, wb, n_ill > 0 ? ctx->logZ2() : nullptr));
-            KL(launch_em_wide(ctx->stream, cnt, D, K, Kg, wb, ctx->sms, &ctx->result()->status));
+            if (!all) KL(launch_em_wide(ctx->stream, cnt, D, K, Kg, wb, ctx->sms, &ctx->result()->status));
             CHECK(prof_end(ctx));
-            KL(launch_reduce_wide(ctx->stream, D, K, Kg, wb, ctx->sms, Nk, S1, S2));
+            if (!all) KL(launch_reduce_wide(ctx->stream, D, K, Kg, wb, ctx->sms, Nk, S1, S2));
             if (n_ill > 0) {
                 double* Nk_c = wb.stats_c;
                 double* S1_c = Nk_c + n_ill;
@@ -650,6 +707,8 @@ int gmm_create(gmm_ctx** out, int device, void* cuda_stream) {
     if (const char* e = std::getenv("GMM_WIDE_MIN_POINTS")) ctx->wide_min_points = std::atof(e);
     if (const char* e = std::getenv("GMM_WIDE_REFINE")) ctx->wide_refine = std::atoi(e) != 0;
     if (const char* e = std::getenv("GMM_WIDE_SPARSE")) ctx->wide_sparse = std::atoi(e);
+    if (const char* e = std::getenv("GMM_WIDE_MODE")) ctx->wide_mode = !std::strcmp(e, "sweeps") ? 1 : !std::strcmp(e, "screen") ? 2 : 0;
+    if (const char* e = std::getenv("GMM_WIDE_PROBE_LIMIT")) ctx->wide_probe_limit = std::atof(e);
     if (const char* e = std::getenv("GMM_WIDE_PIECE")) {
         const long long v = std::atoll(e);
         if (v >= 256 && v <= WIDE_PIECE) ctx->wide_piece = v / 256 * 256;
@@ -742,7 +801,7 @@ int gmm_em_step(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const flo
     DeviceGuard g(ctx->device);
     int path;
     CHECK(ensure_scratch(ctx, D, K));
-    CHECK(prepare_and_choose(ctx, N, D, K, pi, mu, var, &path));
+    CHECK(prepare_and_choose(ctx, N, D, K, pi, mu, var, &path, X, N));
     CHECK(zero_stats(ctx, D, K, Nk, S1, S2, 0));
     CHECK(accumulate_points(ctx, path, X, N, D, K, mu, Nk, S1, S2, 0));
     ctx->last_path = path;
@@ -811,7 +870,7 @@ int gmm_fit(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, float* pi, fl
     int t = 0;
     for (; t < iters; ++t) {
         const int slot = t % LL_SLOTS;
-        CHECK(prepare_and_choose(ctx, N, D, K, pi, mu, var, &path));
+        CHECK(prepare_and_choose(ctx, N, D, K, pi, mu, var, &path, X, N));
         CHECK(zero_stats(ctx, D, K, Nk, S1, S2, slot));
         CHECK(accumulate_points(ctx, path, X, N, D, K, mu, Nk, S1, S2, slot));
         // The update is skipped on the device when the step raised a status bit or left a non-finite log-likelihood

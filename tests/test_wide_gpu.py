@@ -118,21 +118,78 @@ def test_wide_path_with_collapsed_and_low_weight_components(fg, ctx):
 
 
 def test_wide_auto_path_rule(fg, ctx):
-    """AUTO takes the tensor path for D > 128 from 128 points per component on (and K >= 64), the FP32 kernels below; a
-    parameter set in which more than half of the components need exact evaluation runs on the FP32 kernels too."""
+    """AUTO on wide data with K >= 64.  From 128 points per component on: the two tensor sweeps, with a few components
+    evaluated exactly (more than half of them: the FP32 kernels).  Below: one tensor sweep that only screens the pairs, every
+    component evaluated exactly where it matters - unless a sample of the points marks too many pairs (clusters that
+    overlap), in which case the FP32 kernels take the step."""
     rng = np.random.default_rng(5)
     D, K = 256, 64
     assert fg.gmm_auto_path(D, K) == fg.GMM_PATH_TENSOR and fg.gmm_auto_path(D, 32) == fg.GMM_PATH_FP32
     X, pi, mu, var = _clustered(rng, 200 * K, D, K)
     ctx.gmm_set_path(fg.GMM_PATH_AUTO)
     ctx.gmm_em_step(_t(X), _t(pi), _t(mu), _t(var))
-    assert ctx.gmm_last_path() == fg.GMM_PATH_TENSOR
+    assert ctx.gmm_last_path() == fg.GMM_PATH_TENSOR and ctx.gmm_last_exact_count() == 0
     ctx.gmm_em_step(_t(X[:100 * K]), _t(pi), _t(mu), _t(var))
-    assert ctx.gmm_last_path() == fg.GMM_PATH_FP32
+    assert ctx.gmm_last_path() == fg.GMM_PATH_FP32       # (K = 64, D = 256: only 2 marked pairs per point would pay)
+    K2, D2 = 1024, 512
+    X2, pi2, mu2, var2 = _clustered(np.random.default_rng(15), 40 * K2, D2, K2)
+    with fg.Context(0) as c2:
+        _step_and_check(fg, c2, X2, pi2, mu2, var2, "40 points per component: screening sweep + exact pairs")
+        assert c2.gmm_last_path() == fg.GMM_PATH_TENSOR and c2.gmm_last_exact_count() == K2
+        marked, kept, dense = c2.gmm_last_exact_pairs()
+        assert dense == 0 and 40 * K2 <= kept <= marked <= 40 * K2 * 64
     v2 = var.copy()
     v2[:40] = 1e-6
     ctx.gmm_em_step(_t(X), _t(pi), _t(mu), _t(v2))
     assert ctx.gmm_last_path() == fg.GMM_PATH_FP32 and ctx.gmm_last_exact_count() == 0
+    Xo, pio, muo, varo = _clustered(np.random.default_rng(6), 50 * K, D, K, sep=0.01)       # clusters on top of each other
+    _step_and_check(fg, ctx, Xo, pio, muo, varo, "50 points per component, overlapping clusters")
+    assert ctx.gmm_last_path() == fg.GMM_PATH_FP32
+
+
+@pytest.mark.parametrize("N,D,K", [(9_000 + 13, 200, 130), (6_000, 768, 256), (40_000, 320, 96)])
+def test_wide_screen_mode_against_oracle(fg, monkeypatch, N, D, K):
+    """GMM_WIDE_MODE=screen: one tensor sweep screens every (point, component) pair, all marked pairs are evaluated exactly
+    (no component goes through the second tensor sweep).  With collapsed, narrow, light and zero-weight components; pieces
+    of 4096 points; the same bits in a second run."""
+    monkeypatch.setenv("GMM_WIDE_MODE", "screen")
+    monkeypatch.setenv("GMM_WIDE_SPARSE", "2")           # (at these small K the dense kernels would be cheaper: keep to the pairs)
+    monkeypatch.setenv("GMM_WIDE_PIECE", "4096")
+    X, pi, mu, var = _clustered(np.random.default_rng(N + D), N, D, K)
+    mu[0], var[0] = X[7], 1e-6
+    var[1, ::7] = 1e-5
+    pi[2] = 2e-4
+    pi[3] = 0.0
+    pi = (pi / pi.sum()).astype(np.float32)
+    with fg.Context(0) as c:
+        c.gmm_set_path(fg.GMM_PATH_TENSOR)
+        a = _step_and_check(fg, c, X, pi, mu, var, f"screen mode N={N} D={D} K={K}")
+        assert c.gmm_last_path() == fg.GMM_PATH_TENSOR and c.gmm_last_exact_count() == K - 1       # (all with a weight)
+        marked, kept, dense = c.gmm_last_exact_pairs()
+        assert dense == 0 and N <= kept <= marked
+        assert a[0][3] == 0.0
+        Nk, S1, S2, _ = c.gmm_em_step(_t(X), _t(pi), _t(mu), _t(var))
+        for u, v in zip(a, (Nk, S1, S2)):
+            assert np.array_equal(u, v.cpu().numpy())
+
+
+def test_wide_screen_mode_free_running_fit(fg, monkeypatch):
+    monkeypatch.setenv("GMM_WIDE_MODE", "screen")
+    rng = np.random.default_rng(19)
+    N, D, K = 12_000, 256, 64
+    X, pi, mu, var = _clustered(rng, N, D, K)
+    mu0 = X[rng.choice(N, K, replace=False)].copy()
+    var0 = np.tile(X.astype(np.float64).var(0).astype(np.float32), (K, 1))
+    pi0 = np.full(K, 1 / K, np.float32)
+    ref = orc.fit(X, pi0, mu0, var0, 8, var_floor=1e-6)
+    with fg.Context(0) as c:
+        c.gmm_set_path(fg.GMM_PATH_TENSOR)
+        pi_d, mu_d, var_d = _t(pi0), _t(mu0), _t(var0)
+        trace, done = c.gmm_fit(_t(X), pi_d, mu_d, var_d, 8, 1e-6)
+        assert done == 8 and c.gmm_last_path() == fg.GMM_PATH_TENSOR and c.gmm_last_exact_count() > 0
+        np.testing.assert_allclose(trace, ref["trace"], rtol=1e-5)
+        Nk = orc.em_step(X, ref["pi"], ref["mu"], ref["var"])[0]
+        assert np.abs(mu_d.cpu().numpy() - ref["mu"])[Nk >= 1].max() <= 1e-3 * data_scale(X)
 
 
 def test_wide_free_running_fit_matches_the_oracle_trace(fg, ctx):

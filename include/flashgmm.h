@@ -67,19 +67,22 @@ int gmm_destroy(gmm_ctx* ctx);
 /* Select the kernel path for later calls (default GMM_PATH_AUTO).  GMM_EUNSUPPORTED is reported by the compute
  * call, not here, if a forced path cannot run the shape. */
 int gmm_set_path(gmm_ctx* ctx, int path);
-/* 1 if the tensor-core path can run shape (D, K) (D <= 128 and K <= 4096), else 0; GMM_PATH_AUTO uses it whenever
- * this returns 1.  Components too ill-conditioned for the expanded quadratic form (sum_d mu^2 / var beyond what a
- * 22-bit split resolves, e.g. a component collapsed onto one point) have their competitive logits recomputed
- * exactly inside the kernel. */
+/* 1 if a tensor-core path can run shape (D, K) (D <= 1024 and K <= 4096; one kernel design for D <= 128, another for
+ * wider data), else 0.  Components too ill-conditioned for the expanded quadratic form (sum_d mu^2 / var beyond what a
+ * 22-bit split resolves, e.g. a component collapsed onto one point) are evaluated exactly in fp32 where they matter. */
 int gmm_tensor_path_supports(int D, int K);
 /* The path GMM_PATH_AUTO picks for shape (D, K): the tensor-core path when it is supported and the shape fills at
- * least half of a 128-component MMA tile (K >= 64, D >= 8); otherwise the FP32 path, which is both faster and more
- * accurate for small mixtures. */
+ * least half of a 128-component MMA tile (K >= 64, and D >= 8); otherwise the FP32 path, which is both faster and more
+ * accurate for small mixtures.  On wide data (D > 128) a step may still run on the FP32 kernels when the parameters
+ * or the data make that the better choice (more than half of the components ill-conditioned; fewer than 128 points per
+ * component and posteriors too broad for the screening mode): gmm_last_path tells. */
 int gmm_auto_path(int D, int K);
 /* The path (GMM_PATH_FP32 or GMM_PATH_TENSOR) the most recent compute call actually ran. */
 int gmm_last_path(const gmm_ctx* ctx);
 /* How many components the most recent tensor-path step treated as ill-conditioned, i.e. evaluated (where they matter)
- * exactly in fp32 instead of through the expanded quadratic form; 0 after a step on the FP32 path. */
+ * exactly in fp32 instead of through the expanded quadratic form; 0 after a step on the FP32 path.  On wide data
+ * (D > 128) with few points per component the tensor path only screens the (point, component) pairs and evaluates all
+ * that can matter exactly: the count is then the number of components with a positive weight. */
 int gmm_last_exact_count(const gmm_ctx* ctx);
 /* For the most recent tensor-path step on wide data (D > 128) that had such components: how their (point, component)
  * pairs were evaluated.  *marked: pairs the screening sweep could not rule out; *kept: pairs whose exact density came

@@ -1329,11 +1329,13 @@ __device__ __forceinline__ double wide_pair_log2z(const float* __restrict__ xr, 
 // of the final maximum are kept: log-sum-exp into out[i], bit (slot, i) of the transposed map.
 constexpr int CAND_WORDS_PER_LANE = (WIDE_CAND_WORDS + 31) / 32;
 constexpr int CAND_KEEP = 128;
+constexpr int CAND_G = 4;               // marked pairs of a point taken together (their loads overlap)
 __global__ void __launch_bounds__(256) wide_cand_lse_kernel(const float* __restrict__ X, int64_t n, int D, int words,
                                                             const unsigned* __restrict__ cand, unsigned* __restrict__ candT,
                                                             const float* __restrict__ mu_c, const float* __restrict__ w2_c,
                                                             const double* __restrict__ c2d_c, const double* __restrict__ logz,
-                                                            double* __restrict__ out, int* __restrict__ ctl) {
+                                                            double* __restrict__ out, int* __restrict__ ctl,
+                                                            int* __restrict__ slot_cnt) {
     if (ctl[1] != 0) return;
     __shared__ double lbuf[8][CAND_KEEP];
     const int64_t i = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
@@ -1358,19 +1360,94 @@ __global__ void __launch_bounds__(256) wide_cand_lse_kernel(const float* __restr
             if ((wi >> 5) == q) v = bits[q];
         return __shfl_sync(0xffffffffu, v, wi & 31);
     };
+    // exact log2 z of one pair by the whole warp, abandoned once it cannot reach `stop`
+    auto full = [&](int slot, double stop) -> double {
+        return wide_pair_log2z(xr, mu_c + (size_t)slot * D, w2_c + (size_t)slot * D, __ldg(c2d_c + slot), D, lane, stop);
+    };
+    // Most marked pairs are ruled out by their first 128 dimensions.  Those are taken four pairs at a time, one per group
+    // of eight lanes: a lane holds 16 consecutive dimensions of the point (registers) and loads the same 16 of its pair's
+    // component (four 16-byte loads per array), three shuffles sum the group.  (D > 128 on this path.)
+    const int gid = lane >> 3, sub = lane & 7;
+    const bool vec = (D % 4 == 0) && (((reinterpret_cast<uintptr_t>(X) | reinterpret_cast<uintptr_t>(mu_c) | reinterpret_cast<uintptr_t>(w2_c)) & 15) == 0);
+    float xf[16];
+    if (vec) {
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+            const float4 v = __ldg(reinterpret_cast<const float4*>(xr + 16 * sub) + t);
+            xf[4 * t] = v.x; xf[4 * t + 1] = v.y; xf[4 * t + 2] = v.z; xf[4 * t + 3] = v.w;
+        }
+    } else {
+#pragma unroll
+        for (int t = 0; t < 16; ++t) xf[t] = __ldg(xr + 16 * sub + t);
+    }
+    auto first_chunks = [&](const int (&sl)[CAND_G], int cnt, double stop, bool (&alive)[CAND_G]) {
+        const int mine = (gid == 0) ? sl[0] : (gid == 1) ? sl[1] : (gid == 2) ? sl[2] : sl[3];
+        float part = 0.f;
+        if (gid < cnt) {
+            const float* mr = mu_c + (size_t)mine * D + 16 * sub;
+            const float* wr = w2_c + (size_t)mine * D + 16 * sub;
+            if (vec) {
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    const float4 m4 = __ldg(reinterpret_cast<const float4*>(mr) + t);
+                    const float4 w4 = __ldg(reinterpret_cast<const float4*>(wr) + t);
+                    float dd = xf[4 * t] - m4.x;     part = fmaf(dd * dd, w4.x, part);
+                    dd = xf[4 * t + 1] - m4.y;       part = fmaf(dd * dd, w4.y, part);
+                    dd = xf[4 * t + 2] - m4.z;       part = fmaf(dd * dd, w4.z, part);
+                    dd = xf[4 * t + 3] - m4.w;       part = fmaf(dd * dd, w4.w, part);
+                }
+            } else {
+#pragma unroll
+                for (int t = 0; t < 16; ++t) {
+                    const float dd = xf[t] - __ldg(mr + t);
+                    part = fmaf(dd * dd, __ldg(wr + t), part);
+                }
+            }
+        }
+        part += __shfl_xor_sync(0xffffffffu, part, 1);
+        part += __shfl_xor_sync(0xffffffffu, part, 2);
+        part += __shfl_xor_sync(0xffffffffu, part, 4);
+        bool dead = true;
+        if (gid < cnt) {
+            const double c = __ldg(c2d_c + mine);
+            // (the sum of 128 dimensions in another order than the exact evaluation's: a margin of 2 instead of 1)
+            const float room = (stop > -CUDART_INF) ? (float)fmin(fmax(c - stop + 2.0, -3e38), 3e38) : CUDART_INF_F;
+            dead = part > room;
+        }
+        const unsigned am = __ballot_sync(0xffffffffu, !dead && sub == 0);
+#pragma unroll
+        for (int g = 0; g < CAND_G; ++g) alive[g] = ((am >> (8 * g)) & 1u) != 0u;
+    };
     double best = logz[i];
     int idx = 0;
-    for (int wi = 0; wi < words; ++wi) {
-        unsigned word = word_at(wi);
-        while (word) {
-            const int b = __ffs(word) - 1;
-            word &= word - 1;
-            const int slot = wi * 32 + b;
-            const double l = wide_pair_log2z(xr, mu_c + (size_t)slot * D, w2_c + (size_t)slot * D, __ldg(c2d_c + slot), D, lane, best - 40.0);
-            if (idx < CAND_KEEP && lane == 0) lbuf[w][idx] = l;
-            ++idx;
-            if (l > best) best = l;
+    {
+        int sl[CAND_G], cnt = 0;
+        auto flush = [&]() {
+            bool alive[CAND_G];
+            first_chunks(sl, cnt, best - 40.0, alive);
+#pragma unroll
+            for (int g = 0; g < CAND_G; ++g) {
+                if (g < cnt) {
+                    const double l = alive[g] ? full(sl[g], best - 40.0) : -CUDART_INF;
+                    if (idx < CAND_KEEP && lane == 0) lbuf[w][idx] = l;
+                    ++idx;
+                    if (l > best) best = l;
+                }
+            }
+            cnt = 0;
+        };
+        for (int wi = 0; wi < words; ++wi) {
+            unsigned word = word_at(wi);
+            while (word) {
+                const int b = __ffs(word) - 1;
+                word &= word - 1;
+#pragma unroll
+                for (int g = 0; g < CAND_G; ++g)
+                    if (g == cnt) sl[g] = wi * 32 + b;
+                if (++cnt == CAND_G) flush();
+            }
         }
+        if (cnt > 0) flush();
     }
     __syncwarp();
     const double lim = best - 40.0;
@@ -1385,12 +1462,15 @@ __global__ void __launch_bounds__(256) wide_cand_lse_kernel(const float* __restr
             const int slot = wi * 32 + b;
             double l;
             if (idx < CAND_KEEP) l = lbuf[w][idx];
-            else l = wide_pair_log2z(xr, mu_c + (size_t)slot * D, w2_c + (size_t)slot * D, __ldg(c2d_c + slot), D, lane, lim);
+            else l = full(slot, lim);
             ++idx;
             if (l >= lim && l > -CUDART_INF) {               // warp-uniform
                 if (l > m) { ssum = ssum * exp2(m - l) + 1.0; m = l; }
                 else ssum += exp2(l - m);
-                if (lane == 0) atomicOr(candT + (size_t)slot * WIDE_CANDT_WORDS + (i >> 5), 1u << (i & 31));
+                if (lane == 0) {
+                    atomicOr(candT + (size_t)slot * WIDE_CANDT_WORDS + (i >> 5), 1u << (i & 31));
+                    atomicAdd(slot_cnt + slot, 1);
+                }
                 ++kept;
             }
         }
@@ -1408,24 +1488,63 @@ __global__ void __launch_bounds__(256) wide_cand_lse_kernel(const float* __restr
 // thread adds r (x - g), r (x - g)^2 for its dimensions in float64.  The sums are shifted back to the origin and added to
 // the slot's statistics.
 constexpr int MS_CAP = 1024, MS_B = 8;
+constexpr int MS_SEG = WIDE_HEAVY_SEG;     // a component kept for many points of a piece is split over this many blocks ...
+constexpr int MS_SPLIT_MIN = 512;         // ... from this many pairs on
+constexpr int MS_HEAVY = WIDE_HEAVY_SLOTS; // at most this many components are split per piece (the others take one block each)
+
+// Which slots are split: heavy_of[slot] = index of the slot's partial sums or -1, heavy_slot[index] = slot or -1; in slot
+// order, so that nothing depends on timing.  One block of 1024 threads.
+__global__ void __launch_bounds__(1024) wide_heavy_kernel(int n_slots, const int* __restrict__ slot_cnt, int* __restrict__ heavy_of,
+                                                          int* __restrict__ heavy_slot, const int* __restrict__ ctl) {
+    if (ctl[1] != 0) return;
+    __shared__ int wcount[32];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    for (int h = threadIdx.x; h < MS_HEAVY; h += 1024) heavy_slot[h] = -1;
+    __syncthreads();
+    int done = 0;
+    for (int base = 0; base < n_slots; base += 1024) {
+        const int sl = base + threadIdx.x;
+        const bool is = sl < n_slots && slot_cnt[sl] >= MS_SPLIT_MIN;
+        const unsigned b = __ballot_sync(0xffffffffu, is);
+        __syncthreads();
+        if (lane == 0) wcount[w] = __popc(b);
+        __syncthreads();
+        int before = 0, total = 0;
+        for (int j = 0; j < 32; ++j) {
+            if (j < w) before += wcount[j];
+            total += wcount[j];
+        }
+        const int h = done + before + __popc(b & ((1u << lane) - 1u));
+        if (sl < n_slots) heavy_of[sl] = (is && h < MS_HEAVY) ? h : -1;
+        if (is && h < MS_HEAVY) heavy_slot[h] = sl;
+        done += total;
+    }
+}
+
 __global__ void __launch_bounds__(256) wide_cand_mstep_kernel(const float* __restrict__ X, int64_t n, int D, const int* __restrict__ list,
                                                               const unsigned* __restrict__ candT, const float* __restrict__ mu_c,
                                                               const float* __restrict__ w2_c, const double* __restrict__ c2d_c,
                                                               const float* __restrict__ gd, const double* __restrict__ logz_x,
                                                               double* __restrict__ Nk_c, double* __restrict__ S1_c,
-                                                              double* __restrict__ S2_c, const int* __restrict__ ctl) {
+                                                              double* __restrict__ S2_c, const int* __restrict__ ctl,
+                                                              const int* __restrict__ heavy_of, double* __restrict__ heavy_part) {
     if (ctl[1] != 0) return;
-    const int slot = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int slot = blockIdx.x, seg = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (list[slot] < 0) return;
+    const int hv = heavy_of[slot];
+    if (hv < 0 && seg > 0) return;                           // an ordinary slot: one block takes all of its points
     const unsigned* bits = candT + (size_t)slot * WIDE_CANDT_WORDS;
     const int words = (int)((n + 31) >> 5);
-    // thread t owns words [16 t, 16 t + 16): ascending rows across the block
+    // the block's words of the slot's row: all 4096 (16 per thread) or the segment's 512 (2 per thread); thread t owns
+    // consecutive words, so the rows ascend across the block
+    const int wpt = hv < 0 ? 16 : 16 / MS_SEG;
+    const int w0 = (hv < 0 ? 0 : seg * (WIDE_CANDT_WORDS / MS_SEG)) + wpt * tid;
     unsigned mine[16];
     int cnt = 0;
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
-        const int w = 16 * tid + j;
-        mine[j] = (w < words) ? bits[w] : 0u;
+        const int w = w0 + j;
+        mine[j] = (j < wpt && w < words) ? bits[w] : 0u;
         cnt += __popc(mine[j]);
     }
     __shared__ int rows_s[MS_CAP];
@@ -1445,7 +1564,7 @@ __global__ void __launch_bounds__(256) wide_cand_mstep_kernel(const float* __res
         if (j < warp) before += wtot[j];
         total += wtot[j];
     }
-    if (total == 0) return;                                  // block-uniform
+    if (total == 0 && hv < 0) return;                        // block-uniform (a segment still writes its zeros)
     const double c = c2d_c[slot];
     float mu_r[4], w2_r[4], g_r[4];
 #pragma unroll
@@ -1466,7 +1585,7 @@ __global__ void __launch_bounds__(256) wide_cand_mstep_kernel(const float* __res
                 while (word) {
                     const int b = __ffs(word) - 1;
                     word &= word - 1;
-                    if (at >= base && at < base + MS_CAP) rows_s[at - base] = (16 * tid + j) * 32 + b;
+                    if (at >= base && at < base + MS_CAP) rows_s[at - base] = (w0 + j) * 32 + b;
                     ++at;
                 }
             }
@@ -1525,15 +1644,37 @@ __global__ void __launch_bounds__(256) wide_cand_mstep_kernel(const float* __res
         }
         __syncthreads();                                     // rows_s is rewritten by the next pass
     }
-    if (tid == 0) Nk_c[slot] += nk;
+    // sums about the origin: into the slot's statistics, or into the segment's partial sums of a split slot
+    double* oN = hv < 0 ? Nk_c + slot : heavy_part + ((size_t)hv * MS_SEG + seg) * (1 + 2 * (size_t)D);
+    double* o1 = hv < 0 ? S1_c + (size_t)slot * D : oN + 1;
+    double* o2 = hv < 0 ? S2_c + (size_t)slot * D : oN + 1 + D;
+    if (tid == 0) *oN = (hv < 0 ? *oN : 0.0) + nk;
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
         const int d = tid + 256 * q;
         if (d < D) {
             const double g = (double)g_r[q];
-            S1_c[(size_t)slot * D + d] += s1[q] + g * nk;
-            S2_c[(size_t)slot * D + d] += s2[q] + 2.0 * g * s1[q] + g * g * nk;
+            const double a1 = s1[q] + g * nk, a2 = s2[q] + 2.0 * g * s1[q] + g * g * nk;
+            o1[d] = (hv < 0 ? o1[d] : 0.0) + a1;
+            o2[d] = (hv < 0 ? o2[d] : 0.0) + a2;
         }
+    }
+}
+
+// The split slots' statistics: their segments' partial sums in order.
+__global__ void __launch_bounds__(256) wide_heavy_combine_kernel(int D, const int* __restrict__ heavy_slot, const double* __restrict__ heavy_part,
+                                                                 double* __restrict__ Nk_c, double* __restrict__ S1_c,
+                                                                 double* __restrict__ S2_c, const int* __restrict__ ctl) {
+    if (ctl[1] != 0) return;
+    const int slot = heavy_slot[blockIdx.x];
+    if (slot < 0) return;
+    const double* p = heavy_part + (size_t)blockIdx.x * MS_SEG * (1 + 2 * (size_t)D);
+    for (int e = threadIdx.x; e < 1 + 2 * D; e += 256) {
+        double s = 0.0;
+        for (int g = 0; g < MS_SEG; ++g) s += p[(size_t)g * (1 + 2 * (size_t)D) + e];
+        if (e == 0) Nk_c[slot] += s;
+        else if (e <= D) S1_c[(size_t)slot * D + (e - 1)] += s;
+        else S2_c[(size_t)slot * D + (e - 1 - D)] += s;
     }
 }
 
@@ -1808,6 +1949,7 @@ cudaError_t launch_cand_clear_wide(cudaStream_t s, int64_t n, int n_slots, const
     cudaError_t e = cudaMemsetAsync(wb.ctl, 0, 8 * sizeof(int), s);
     if (e == cudaSuccess) e = cudaMemsetAsync(wb.cand, 0, (size_t)n * words * sizeof(unsigned), s);
     if (e == cudaSuccess) e = cudaMemsetAsync(wb.candT, 0, (size_t)n_slots * WIDE_CANDT_WORDS * sizeof(unsigned), s);
+    if (e == cudaSuccess) e = cudaMemsetAsync(wb.slot_cnt, 0, (size_t)n_slots * sizeof(int), s);
     return e;
 }
 
@@ -1825,7 +1967,7 @@ cudaError_t launch_cand_lse_wide(cudaStream_t s, const float* X, int64_t n, int 
                                  double* logz_ill) {
     const int words = (n_slots + 31) / 32;
     wide_cand_lse_kernel<<<(unsigned)((n + 7) / 8), 256, 0, s>>>(X, n, D, words, wb.cand, wb.candT, wb.mu_c, wb.w2_c, wb.c2d_c, wb.logz,
-                                                                 logz_ill, wb.ctl);
+                                                                 logz_ill, wb.ctl, wb.slot_cnt);
     return cudaGetLastError();
 }
 
@@ -1833,8 +1975,14 @@ cudaError_t launch_cand_mstep_wide(cudaStream_t s, const float* X, int64_t n, in
     double* Nk_c = wb.stats_c;
     double* S1_c = Nk_c + n_slots;
     double* S2_c = S1_c + (size_t)n_slots * D;
-    wide_cand_mstep_kernel<<<(unsigned)n_slots, 256, 0, s>>>(X, n, D, wb.ill_list, wb.candT, wb.mu_c, wb.w2_c, wb.c2d_c, wb.gd,
-                                                             wb.logz_x, Nk_c, S1_c, S2_c, wb.ctl);
+    wide_heavy_kernel<<<1, 1024, 0, s>>>(n_slots, wb.slot_cnt, wb.heavy_of, wb.heavy_slot, wb.ctl);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    wide_cand_mstep_kernel<<<dim3((unsigned)n_slots, MS_SEG), 256, 0, s>>>(X, n, D, wb.ill_list, wb.candT, wb.mu_c, wb.w2_c, wb.c2d_c, wb.gd,
+                                                                        wb.logz_x, Nk_c, S1_c, S2_c, wb.ctl, wb.heavy_of, wb.heavy_part);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    wide_heavy_combine_kernel<<<MS_HEAVY, 256, 0, s>>>(D, wb.heavy_slot, wb.heavy_part, Nk_c, S1_c, S2_c, wb.ctl);
     return cudaGetLastError();
 }
 

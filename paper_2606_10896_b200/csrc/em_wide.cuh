@@ -15,6 +15,7 @@ constexpr int WIDE_TILE = 128;               // points per tile of the first swe
 constexpr int WIDE_MAX_ILL = WIDE_MAX_K + 64; // slots of the list of components evaluated exactly (all of them may be; + the gap)
 constexpr int WIDE_LL_BLOCKS = 64;           // per-block partial sums of the log-likelihood
 constexpr int WIDE_MAX_TOP = 10;             // candidates per point sweep 1 can report (the top-m assignment asks for m + 2)
+constexpr int WIDE_HEAVY_SLOTS = 256, WIDE_HEAVY_SEG = 8;    // see wide_cand_mstep_kernel
 constexpr int WIDE_CAND_WORDS = (WIDE_MAX_ILL + 31) / 32;   // 32-bit words of a point's row of the candidate bitmap, at most
 constexpr int WIDE_CANDT_WORDS = (int)(WIDE_PIECE / 32);    // words of a slot's row of the transposed bitmap
 
@@ -68,6 +69,10 @@ struct WideBuffers {
     float* n2;      // [WIDE_PIECE] |x_i - g|^2
     unsigned* cand; // [WIDE_PIECE][words] bit (i, slot): the pair may matter (set by sweep 1)
     unsigned* candT;// [WIDE_MAX_ILL][WIDE_CANDT_WORDS] bit (slot, i): the pair matters (set by the exact evaluation)
+    int* slot_cnt;  // [slots] pairs kept per slot in the current piece
+    int* heavy_of;  // [slots] index of a slot's partial sums when its points are split over several blocks, else -1
+    int* heavy_slot;// [WIDE_HEAVY_SLOTS] the slot of each set of partial sums, -1 if unused
+    double* heavy_part;    // [WIDE_HEAVY_SLOTS][WIDE_HEAVY_SEG][1 + 2 D] partial (N_k, S1, S2) of the split slots' segments
     int* ctl;       // [8]: [0] pairs sweep 1 let through, [1] nonzero: too many, the FP32 kernels evaluate the sub-mixture
                     //      densely, [2] nonzero: the pairs are evaluated one by one, [3] pairs that mattered
 };

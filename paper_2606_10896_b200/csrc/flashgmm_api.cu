@@ -34,7 +34,7 @@ struct ScratchLayout {
     size_t tc_phi, tc_plo, tc_tk, tc_ck, tc_sd, tc_kap, tc_gd, tc_illb, tc_flags, tc_xg, tc_xl, tc_partial, tc_llpart, tc_partial_bytes, tc_yhi, tc_ylo, tc_phirm, tc_plorm, tc_tkck, tc_illlist, tc_illcache, tc_decdim, tc_decw, tc_decmu;
     bool tc;
     // the tensor-core path for D > 128
-    size_t w_sd, w_kap, w_gd, w_phi, w_plo, w_tk, w_tkck, w_ckd, w_cref, w_illb, w_flags, w_yhi, w_ylo, w_logz, w_partial, w_llpart, w_illlist, w_muc, w_w2c, w_c2dc, w_statsc, w_top, w_logzx, w_compof, w_scra, w_scrw, w_scr, w_slotof, w_scrmask, w_n2, w_cand, w_candT, w_ctl, w_scre;
+    size_t w_sd, w_kap, w_gd, w_phi, w_plo, w_tk, w_tkck, w_ckd, w_cref, w_illb, w_flags, w_yhi, w_ylo, w_logz, w_partial, w_llpart, w_illlist, w_muc, w_w2c, w_c2dc, w_statsc, w_top, w_logzx, w_compof, w_scra, w_scrw, w_scr, w_slotof, w_scrmask, w_n2, w_cand, w_candT, w_ctl, w_scre, w_slotcnt, w_heavyof, w_heavyslot, w_heavypart;
     size_t w_partial_bytes;
     bool wide;
 };
@@ -89,7 +89,7 @@ ScratchLayout scratch_layout(int D, int K, bool planes) {
         L.tc_ylo = take(TC_YPLANE_BYTES);
     }
     L.w_sd = L.w_kap = L.w_gd = L.w_phi = L.w_plo = L.w_tk = L.w_tkck = L.w_ckd = L.w_cref = L.w_illb = L.w_flags = L.w_yhi = L.w_ylo = L.w_logz = L.w_partial = L.w_llpart = L.w_illlist = L.w_muc = L.w_w2c = L.w_c2dc = L.w_statsc = L.w_top = L.w_logzx = 0;
-    L.w_compof = L.w_scra = L.w_scrw = L.w_scr = L.w_slotof = L.w_scrmask = L.w_n2 = L.w_cand = L.w_candT = L.w_ctl = L.w_scre = 0;
+    L.w_compof = L.w_scra = L.w_scrw = L.w_scr = L.w_slotof = L.w_scrmask = L.w_n2 = L.w_cand = L.w_candT = L.w_ctl = L.w_scre = L.w_slotcnt = L.w_heavyof = L.w_heavyslot = L.w_heavypart = 0;
     L.w_partial_bytes = 0;
     L.wide = wide_supports(D, K) && planes;
     if (L.wide) {
@@ -117,6 +117,10 @@ ScratchLayout scratch_layout(int D, int K, bool planes) {
         L.w_candT = take(slots * WIDE_CANDT_WORDS * 4);
         L.w_ctl = take(32);
         L.w_scre = take((size_t)wp.rows * 4);
+        L.w_slotcnt = take(slots * 4);
+        L.w_heavyof = take(slots * 4);
+        L.w_heavyslot = take((size_t)WIDE_HEAVY_SLOTS * 4);
+        L.w_heavypart = take((size_t)WIDE_HEAVY_SLOTS * WIDE_HEAVY_SEG * (1 + 2 * (size_t)D) * 8);
         L.w_logz = take((size_t)WIDE_PIECE * 8);
         L.w_top = take((size_t)WIDE_PIECE * 2 * WIDE_MAX_TOP * 4);
         L.w_logzx = take((size_t)WIDE_PIECE * 8);
@@ -270,6 +274,10 @@ struct gmm_ctx {
         b.candT = reinterpret_cast<unsigned*>(scratch + lay.w_candT);
         b.ctl = reinterpret_cast<int*>(scratch + lay.w_ctl);
         b.scr_e = reinterpret_cast<float*>(scratch + lay.w_scre);
+        b.slot_cnt = reinterpret_cast<int*>(scratch + lay.w_slotcnt);
+        b.heavy_of = reinterpret_cast<int*>(scratch + lay.w_heavyof);
+        b.heavy_slot = reinterpret_cast<int*>(scratch + lay.w_heavyslot);
+        b.heavy_part = reinterpret_cast<double*>(scratch + lay.w_heavypart);
         return b;
     }
 };
@@ -579,7 +587,10 @@ int accumulate_points(gmm_ctx* ctx, int path, const float* X, int64_t n, int D, 
                 double* Nk_c = wb.stats_c;
                 double* S1_c = Nk_c + n_ill;
                 double* S2_c = S1_c + (size_t)n_ill * D;
-                if (screen) KL(launch_cand_mstep_wide(ctx->stream, Xs, cnt, D, n_ill, wb));
+                if (screen) {
+                    KL(launch_cand_mstep_wide(ctx->stream, Xs, cnt, D, n_ill, wb));
+                    ctx->launches += 2;
+                }
                 if (n_a > 0) {
                     KL(launch_mstep_fp32(ctx->stream, Xs, cnt, D, n_a, wb.mu_c, wb.w2_c, wb.c2d_c, ctx->center(), wb.logz_x, ctx->partials(), plan_a, true, dense_if));
                     KL(launch_reduce_partials(ctx->stream, D, n_a, plan_a.splits, ctx->partials(), ctx->center(), Nk_c, S1_c, S2_c, true));

@@ -1328,7 +1328,8 @@ __device__ __forceinline__ double wide_pair_log2z(const float* __restrict__ xr, 
 // components to begin with: logz); the first 128 values are kept in shared memory.  Second round: the pairs within 2^-40
 // of the final maximum are kept: log-sum-exp into out[i], bit (slot, i) of the transposed map.
 constexpr int CAND_WORDS_PER_LANE = (WIDE_CAND_WORDS + 31) / 32;
-constexpr int CAND_KEEP = 128;
+constexpr int CAND_KEEP = 256;          // exact values of a point's first pairs kept between the two rounds
+constexpr int CAND_LIST = 256;          // marked slots of a point listed in shared memory (more: the row is scanned instead)
 constexpr int CAND_G = 4;               // marked pairs of a point taken together (their loads overlap)
 __global__ void __launch_bounds__(256) wide_cand_lse_kernel(const float* __restrict__ X, int64_t n, int D, int words,
                                                             const unsigned* __restrict__ cand, unsigned* __restrict__ candT,
@@ -1338,6 +1339,7 @@ __global__ void __launch_bounds__(256) wide_cand_lse_kernel(const float* __restr
                                                             int* __restrict__ slot_cnt) {
     if (ctl[1] != 0) return;
     __shared__ double lbuf[8][CAND_KEEP];
+    __shared__ unsigned short slist[8][CAND_LIST];
     const int64_t i = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     if (i >= n) return;
@@ -1361,14 +1363,54 @@ __global__ void __launch_bounds__(256) wide_cand_lse_kernel(const float* __restr
         return __shfl_sync(0xffffffffu, v, wi & 31);
     };
     // exact log2 z of one pair by the whole warp, abandoned once it cannot reach `stop`
+    // (With rows of whole 16-byte groups the point stays in registers, a lane holding dimensions 4 l .. 4 l + 3 of every
+    // 128, and a component's row comes in 16-byte loads: a quarter of the instructions of the general routine.  A lane
+    // sums its 4 dimensions of each 128 in fp32, the chunk sums are added in float64, fixed butterfly at the end; the
+    // running total is looked at after the first 128 dimensions and then after every 256.)
+    const bool vec = (D % 4 == 0) && (((reinterpret_cast<uintptr_t>(X) | reinterpret_cast<uintptr_t>(mu_c) | reinterpret_cast<uintptr_t>(w2_c)) & 15) == 0);
+    float4 xq[8];
+    if (vec) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+            xq[j] = (128 * j + 4 * lane < D) ? __ldg(reinterpret_cast<const float4*>(xr + 128 * j) + lane) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
     auto full = [&](int slot, double stop) -> double {
-        return wide_pair_log2z(xr, mu_c + (size_t)slot * D, w2_c + (size_t)slot * D, __ldg(c2d_c + slot), D, lane, stop);
+        const double c = __ldg(c2d_c + slot);
+        if (!vec) return wide_pair_log2z(xr, mu_c + (size_t)slot * D, w2_c + (size_t)slot * D, c, D, lane, stop);
+        const float4* mr = reinterpret_cast<const float4*>(mu_c + (size_t)slot * D) + lane;
+        const float4* wr = reinterpret_cast<const float4*>(w2_c + (size_t)slot * D) + lane;
+        const float room = (stop > -CUDART_INF) ? (float)fmin(fmax(c - stop + 1.0, -3e38), 3e38) : CUDART_INF_F;
+        double q = 0.0;
+        float run = 0.f;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            if (128 * j < D) {                               // warp-uniform
+                float part = 0.f;
+                if (128 * j + 4 * lane < D) {
+                    const float4 m4 = __ldg(mr + 32 * j), w4 = __ldg(wr + 32 * j);
+                    float dd = xq[j].x - m4.x;  part = fmaf(dd * dd, w4.x, part);
+                    dd = xq[j].y - m4.y;        part = fmaf(dd * dd, w4.y, part);
+                    dd = xq[j].z - m4.z;        part = fmaf(dd * dd, w4.z, part);
+                    dd = xq[j].w - m4.w;        part = fmaf(dd * dd, w4.w, part);
+                }
+                q += (double)part;
+                run += part;
+                if (j == 0 || (j & 1) == 0) {                // after 128 dimensions, then after every 256
+                    float tot = run;
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, o);
+                    if (tot > room) return -CUDART_INF;
+                }
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
+        return c - q;
     };
     // Most marked pairs are ruled out by their first 128 dimensions.  Those are taken four pairs at a time, one per group
     // of eight lanes: a lane holds 16 consecutive dimensions of the point (registers) and loads the same 16 of its pair's
     // component (four 16-byte loads per array), three shuffles sum the group.  (D > 128 on this path.)
     const int gid = lane >> 3, sub = lane & 7;
-    const bool vec = (D % 4 == 0) && (((reinterpret_cast<uintptr_t>(X) | reinterpret_cast<uintptr_t>(mu_c) | reinterpret_cast<uintptr_t>(w2_c)) & 15) == 0);
     float xf[16];
     if (vec) {
 #pragma unroll
@@ -1418,6 +1460,34 @@ __global__ void __launch_bounds__(256) wide_cand_lse_kernel(const float* __restr
 #pragma unroll
         for (int g = 0; g < CAND_G; ++g) alive[g] = ((am >> (8 * g)) & 1u) != 0u;
     };
+    // The point's marked slots, in ascending order, as a list in shared memory (scanning the 130 words of the row twice
+    // cost more than evaluating the pairs): word lane + 32 q belongs to lane `lane`, so the order is (q, lane, bit).
+    int total = 0;
+    {
+        int base = 0;
+#pragma unroll
+        for (int q = 0; q < CAND_WORDS_PER_LANE; ++q) {
+            const int c = __popc(bits[q]);
+            int incl = c;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int t = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += t;
+            }
+            int at = base + incl - c;
+            unsigned word = bits[q];
+            while (word) {
+                const int b = __ffs(word) - 1;
+                word &= word - 1;
+                if (at < CAND_LIST) slist[w][at] = (unsigned short)((lane + 32 * q) * 32 + b);
+                ++at;
+            }
+            base += __shfl_sync(0xffffffffu, incl, 31);
+        }
+        total = base;
+    }
+    __syncwarp();
+    const bool listed = total <= CAND_LIST;                   // (else: the row is scanned word by word, as a fallback)
     double best = logz[i];
     int idx = 0;
     {
@@ -1436,42 +1506,57 @@ __global__ void __launch_bounds__(256) wide_cand_lse_kernel(const float* __restr
             }
             cnt = 0;
         };
-        for (int wi = 0; wi < words; ++wi) {
-            unsigned word = word_at(wi);
-            while (word) {
-                const int b = __ffs(word) - 1;
-                word &= word - 1;
+        if (listed) {
+            for (int e = 0; e < total; e += CAND_G) {
+                cnt = (total - e < CAND_G) ? (total - e) : CAND_G;
 #pragma unroll
-                for (int g = 0; g < CAND_G; ++g)
-                    if (g == cnt) sl[g] = wi * 32 + b;
-                if (++cnt == CAND_G) flush();
+                for (int g = 0; g < CAND_G; ++g) sl[g] = (g < cnt) ? (int)slist[w][e + g] : 0;
+                flush();
             }
+        } else {
+            for (int wi = 0; wi < words; ++wi) {
+                unsigned word = word_at(wi);
+                while (word) {
+                    const int b = __ffs(word) - 1;
+                    word &= word - 1;
+#pragma unroll
+                    for (int g = 0; g < CAND_G; ++g)
+                        if (g == cnt) sl[g] = wi * 32 + b;
+                    if (++cnt == CAND_G) flush();
+                }
+            }
+            if (cnt > 0) flush();
         }
-        if (cnt > 0) flush();
     }
     __syncwarp();
     const double lim = best - 40.0;
     double m = -CUDART_INF, ssum = 0.0;
     int kept = 0;
-    idx = 0;
-    for (int wi = 0; wi < words; ++wi) {
-        unsigned word = word_at(wi);
-        while (word) {
-            const int b = __ffs(word) - 1;
-            word &= word - 1;
-            const int slot = wi * 32 + b;
-            double l;
-            if (idx < CAND_KEEP) l = lbuf[w][idx];
-            else l = full(slot, lim);
-            ++idx;
-            if (l >= lim && l > -CUDART_INF) {               // warp-uniform
-                if (l > m) { ssum = ssum * exp2(m - l) + 1.0; m = l; }
-                else ssum += exp2(l - m);
-                if (lane == 0) {
-                    atomicOr(candT + (size_t)slot * WIDE_CANDT_WORDS + (i >> 5), 1u << (i & 31));
-                    atomicAdd(slot_cnt + slot, 1);
-                }
-                ++kept;
+    auto second = [&](int slot, int at) {
+        double l;
+        if (at < CAND_KEEP) l = lbuf[w][at];
+        else l = full(slot, lim);
+        if (l >= lim && l > -CUDART_INF) {                   // warp-uniform
+            if (l > m) { ssum = ssum * exp2(m - l) + 1.0; m = l; }
+            else ssum += exp2(l - m);
+            if (lane == 0) {
+                atomicOr(candT + (size_t)slot * WIDE_CANDT_WORDS + (i >> 5), 1u << (i & 31));
+                atomicAdd(slot_cnt + slot, 1);
+            }
+            ++kept;
+        }
+    };
+    if (listed) {
+        for (int e = 0; e < total; ++e) second((int)slist[w][e], e);
+    } else {
+        idx = 0;
+        for (int wi = 0; wi < words; ++wi) {
+            unsigned word = word_at(wi);
+            while (word) {
+                const int b = __ffs(word) - 1;
+                word &= word - 1;
+                second(wi * 32 + b, idx);
+                ++idx;
             }
         }
     }

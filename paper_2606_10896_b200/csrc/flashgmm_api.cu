@@ -179,7 +179,7 @@ struct gmm_ctx {
     int wide_mode = 0;               // GMM_WIDE_MODE: 0 = automatic, 1 = "sweeps" (two tensor sweeps, few components exact),
                                      // 2 = "screen" (one tensor sweep screens every pair, every component evaluated exactly)
     double wide_probe_limit = 0.0;   // automatic mode: "screen" while a sample of the points has at most this many marked pairs per
-                                     // point (0: K D / 8192)
+                                     // point (0: K D / 70000, or K D / 8192 below 128 points per component)
     bool wide_screen_all = false;    // the current step runs in "screen" mode
     int wide_sparse = 1;             // GMM_WIDE_SPARSE: 0 = the listed components always go through the dense FP32 kernels,
                                      // 1 = pair by pair unless sweep 1 marks too many pairs, 2 = always pair by pair (tests)
@@ -440,12 +440,16 @@ int prepare_and_choose(gmm_ctx* ctx, int64_t N, int D, int K, const float* pi, c
         const WideBuffers wb = ctx->wide();
         int fl[8];
         const bool can_probe = Xprobe != nullptr && n_probe >= 1;
-        // Automatic choice: "sweeps" from 128 points per component on (measured at config 5's shape, steady state: 105 ms per
-        // million points against 142 for "screen", whose exact evaluation of 26 marked pairs per point costs more than the
-        // second sweep); "screen" below that, where "sweeps" would find most components light and the alternative is the FP32
-        // kernels (1580 ms per million points) - provided a sample of the points marks few enough pairs.
+        // Automatic choice, step by step: the screening sweep is tried on the first 8192 rows, and "screen" is taken if it marks
+        // few enough pairs per point.  A marked pair costs about 1.3 ns (exact evaluation) and a kept one 5 ns more (its
+        // statistics); what "screen" saves is the second tensor sweep, K D / 50 ps per point (60 ns at config 5's shape), so
+        // from 128 points per component on the limit is K D / 70000 marked pairs per point - config 5: 45, which its first
+        // three iterations from a data-row initialisation exceed (74, 97, 71 at N = 1M: 180-300 ms per million points
+        // against 122 for "sweeps") and the later ones do not (26 at N = 1M: 82 ms against 101; 37-42 at N = 10M: 89-96
+        // against 105).  Below 128 points per component "sweeps" is no
+        // alternative (it would list most components as light) and the FP32 kernels cost K D / 2 ns per point: K D / 8192.
         const bool few_points = N < WIDE_AUTO_MIN_POINTS_PER_COMPONENT * K;
-        if (ctx->wide_mode == 2 || (ctx->wide_mode == 0 && can_probe && few_points)) {
+        if (ctx->wide_mode == 2 || (ctx->wide_mode == 0 && can_probe)) {
             KL(launch_prepare_wide(ctx->stream, D, K, pi, mu, var, wb, limit, INFINITY));      // every component is listed
             ctx->launches += 4;
             CU(cudaMemcpyAsync(fl, wb.flags, sizeof(fl), cudaMemcpyDeviceToHost, ctx->stream));
@@ -463,9 +467,8 @@ int prepare_and_choose(gmm_ctx* ctx, int64_t N, int D, int K, const float* pi, c
                 int marks = 0;
                 CU(cudaMemcpyAsync(&marks, wb.ctl, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
                 CU(cudaStreamSynchronize(ctx->stream));
-                // (a marked pair costs about 1.3 ns, mostly for being ruled out after its first 128 dimensions; the FP32 kernels
-                // cost K D / 2000 ns per point: the pair route is taken while it is clearly the cheaper one)
-                ok = (double)marks <= (ctx->wide_probe_limit > 0.0 ? ctx->wide_probe_limit : (double)n_list * D / 8192.0) * (double)np;
+                const double auto_limit = (double)n_list * D / (few_points ? 8192.0 : 70000.0);
+                ok = (double)marks <= (ctx->wide_probe_limit > 0.0 ? ctx->wide_probe_limit : auto_limit) * (double)np;
             }
             if (ok) {
                 ctx->wide_n_ill = fl[4];

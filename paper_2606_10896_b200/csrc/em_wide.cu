@@ -1331,7 +1331,7 @@ constexpr int CAND_WORDS_PER_LANE = (WIDE_CAND_WORDS + 31) / 32;
 constexpr int CAND_KEEP = 256;          // exact values of a point's first pairs kept between the two rounds
 constexpr int CAND_LIST = 256;          // marked slots of a point listed in shared memory (more: the row is scanned instead)
 constexpr int CAND_G = 4;               // marked pairs of a point taken together (their loads overlap)
-__global__ void __launch_bounds__(256) wide_cand_lse_kernel(const float* __restrict__ X, int64_t n, int D, int words,
+__global__ void __launch_bounds__(256, 4) wide_cand_lse_kernel(const float* __restrict__ X, int64_t n, int D, int words,
                                                             const unsigned* __restrict__ cand, unsigned* __restrict__ candT,
                                                             const float* __restrict__ mu_c, const float* __restrict__ w2_c,
                                                             const double* __restrict__ c2d_c, const double* __restrict__ logz,

@@ -584,7 +584,6 @@ int accumulate_points(gmm_ctx* ctx, int path, const float* X, int64_t n, int D, 
             }
             KL(launch_merge_ll_wide(ctx->stream, cnt, wb, n_ill > 0 ? ctx->logZ2() : nullptr));
             if (!all) KL(launch_em_wide(ctx->stream, cnt, D, K, Kg, wb, ctx->sms, &ctx->result()->status));
-            CHECK(prof_end(ctx));
             if (!all) KL(launch_reduce_wide(ctx->stream, D, K, Kg, wb, ctx->sms, Nk, S1, S2));
             if (n_ill > 0) {
                 double* Nk_c = wb.stats_c;
@@ -605,6 +604,7 @@ int accumulate_points(gmm_ctx* ctx, int path, const float* X, int64_t n, int D, 
                 }
                 if (screen) KL(launch_cand_count_wide(ctx->stream, wb));
             }
+            CHECK(prof_end(ctx));                             // (the bracket holds every kernel of the piece)
         }
         if (n_ill > 0) KL(launch_ill_scatter_wide(ctx->stream, D, K, n_ill, wb, Nk, S1, S2));
         KL(launch_reduce_ll(ctx->stream, wb.llpart, WIDE_LL_BLOCKS, &ctx->result()->ll[slot], true));

@@ -22,8 +22,15 @@
 // Precision as on the D <= 128 path (every operand split into two fp16 values; three products per contraction), with
 // kap_d chosen so that a component's own points give terms of zero mean in every dimension: the accumulators then stay
 // small (tens, not D / 2), and with them the truncation error of the tensor core's fp32 accumulation.
-// Ill-conditioned components (error estimate above the limit) are not handled here: the host sends such parameter
-// sets to the FP32 kernels.
+//
+// Components the expanded form cannot carry (collapsed or narrow ones, and ones that hold few points) are "listed": they
+// sit behind the others in the order the sweeps see the components, sweep 2 leaves them out, and sweep 1 only SCREENS
+// them - it marks, in a bitmap, the (point, component) pairs whose approximate log2 z plus a rigorous error bound can
+// come within 2^-40 of the point's best.  The marked pairs are then evaluated exactly in fp32, pair by pair
+// (wide_cand_lse_kernel, wide_cand_mstep_kernel), or, when they are too many, densely by the FP32 kernels.  In the
+// "screen" mode EVERY component is listed: one tensor sweep decides which pairs are looked at, all statistics come from
+// exact evaluations.  The same screening, with the candidates ranked by upper bounds, gives the top-m assignment
+// (wide_assign_refine_kernel).
 #include "internal.cuh"
 #include "em_tc.cuh"
 #include "em_wide.cuh"
@@ -73,6 +80,7 @@ struct LseParams {
     unsigned* cand;      // [n][cand_words]
     int cand_words;
     int scr_group;       // first group of 256 columns that holds listed components (they hold nothing else from there on)
+    int hi_group;        // from this group on only the leading product (Y_hi P_hi) is formed: screening with wider allowances
     int* ctl;
 };
 
@@ -161,6 +169,7 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
             for (int g = 0; g < NG; ++g) {
                 const int nch = (NC - 2 * g < 2) ? (NC - 2 * g) : 2;
                 const bool screening = p.screen && g >= p.scr_group;
+                const bool hi_grp = g >= p.hi_group;          // (only screening groups are ever of this kind)
                 if (screening) {
                     // What a pair is screened against: the point's maximum over the evaluated components (final by now; the
                     // two warpgroups merge theirs at the first screening group) and the largest LOWER bound among the listed
@@ -205,8 +214,10 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
                                         const float4 q = __ldg(tc4 + (j >> 1));
                                         const float4 sq = __ldg(sc4 + (j >> 1));
                                         const float2 se = __ldg(se2 + (j >> 1));
-                                        const float u0 = fmaf(__uint_as_float(v[j]) + __uint_as_float(vc[j]), q.x, fmaf(sq.y, nrm, sq.x));
-                                        const float u1 = fmaf(__uint_as_float(v[j + 1]) + __uint_as_float(vc[j + 1]), q.z, fmaf(sq.w, nrm, sq.z));
+                                        const float a0 = hi_grp ? __uint_as_float(v[j]) : __uint_as_float(v[j]) + __uint_as_float(vc[j]);
+                                        const float a1 = hi_grp ? __uint_as_float(v[j + 1]) : __uint_as_float(v[j + 1]) + __uint_as_float(vc[j + 1]);
+                                        const float u0 = fmaf(a0, q.x, fmaf(sq.y, nrm, sq.x));
+                                        const float u1 = fmaf(a1, q.z, fmaf(sq.w, nrm, sq.z));
                                         // lower bounds: the upper bound minus twice the allowance (fmaxf drops a NaN)
                                         thr_base = fmaxf(thr_base, fmaxf(u0 - 2.f * fmaf(sq.y, nrm, se.x), u1 - 2.f * fmaf(sq.w, nrm, se.y)));
                                         const float thr = thr_base - 40.f;
@@ -311,7 +322,7 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
         int64_t g = 0;
         bool ok = true;
         const uint64_t pol_keep = l2_policy_evict_last(), pol_stream = l2_policy_evict_first();
-        auto item = [&](const CUtensorMap* mh, const CUtensorMap* ml, int32_t row, int32_t z, bool keep) -> bool {
+        auto item = [&](const CUtensorMap* mh, const CUtensorMap* ml, int32_t row, int32_t z, bool keep, bool hi_only) -> bool {
             const int slot = (int)(g % L_SLOTS);
             const int64_t use = g / L_SLOTS;
             if (use > 0) {
@@ -321,10 +332,10 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
             }
             if (elect_one()) {
                 const uint32_t dst = smem_u32(smem + slot * SLOT);
-                bar_expect_tx(BAR(LB_FULL + slot), SLOT);
+                bar_expect_tx(BAR(LB_FULL + slot), hi_only ? SLOT / 2 : SLOT);
                 // the coefficient atoms are read by every CTA for every tile, the tile's own atoms once
                 tma_load_3d_hint(dst, mh, 0, row, z, BAR(LB_FULL + slot), keep ? pol_keep : pol_stream);
-                tma_load_3d_hint(dst + SLOT / 2, ml, 0, row, z, BAR(LB_FULL + slot), keep ? pol_keep : pol_stream);
+                if (!hi_only) tma_load_3d_hint(dst + SLOT / 2, ml, 0, row, z, BAR(LB_FULL + slot), keep ? pol_keep : pol_stream);
             }
             __syncwarp();
             ++g;
@@ -335,8 +346,9 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
             for (int gq = 0; gq < NG && ok; ++gq) {
                 const int nch = (NC - 2 * gq < 2) ? (NC - 2 * gq) : 2;
                 for (int z = 0; z < NZ && ok; ++z) {
-                    ok = item(&tm_yhi, &tm_ylo, row0, z, false);
-                    for (int c = 0; c < nch && ok; ++c) ok = item(&tm_phi, &tm_plo, (2 * gq + c) * 128, z, true);
+                    const bool hi_only = gq >= p.hi_group;
+                    ok = item(&tm_yhi, &tm_ylo, row0, z, false, hi_only);
+                    for (int c = 0; c < nch && ok; ++c) ok = item(&tm_phi, &tm_plo, (2 * gq + c) * 128, z, true, hi_only);
                 }
             }
         }
@@ -379,10 +391,12 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
                             const uint32_t d = tmem + c * 128, dc = tmem + 256 + c * 128;
                             // the two small cross products into their own accumulator, the leading product into the main one:
                             // the same three chains, in the same order, as the E-step of sweep 2
+                            if (gq < p.hi_group) {
 #pragma unroll
-                            for (int j = 0; j < 4; ++j) mma_ss(dc, ah + ((j * 32) >> 4), bl + ((j * 32) >> 4), idesc, (z > 0 || j > 0) ? 1u : 0u);
+                                for (int j = 0; j < 4; ++j) mma_ss(dc, ah + ((j * 32) >> 4), bl + ((j * 32) >> 4), idesc, (z > 0 || j > 0) ? 1u : 0u);
 #pragma unroll
-                            for (int j = 0; j < 4; ++j) mma_ss(dc, al + ((j * 32) >> 4), bh + ((j * 32) >> 4), idesc, 1u);
+                                for (int j = 0; j < 4; ++j) mma_ss(dc, al + ((j * 32) >> 4), bh + ((j * 32) >> 4), idesc, 1u);
+                            }
 #pragma unroll
                             for (int j = 0; j < 4; ++j) mma_ss(d, ah + ((j * 32) >> 4), bh + ((j * 32) >> 4), idesc, (z > 0 || j > 0) ? 1u : 0u);
                             mma_commit(BAR(LB_EMPTY + sp));
@@ -895,6 +909,7 @@ __global__ void __launch_bounds__(256) wide_flag_kernel(int D, int Dpad, int K, 
                                                         const float* __restrict__ sd, const float* __restrict__ kap,
                                                         const float* __restrict__ gd, float* __restrict__ illb,
                                                         float* __restrict__ scra, float* __restrict__ scrw,
+                                                        float* __restrict__ scra_hi, float* __restrict__ scrw_hi,
                                                         float cond_limit, float min_weight, int* __restrict__ flags) {
     __shared__ double red[4][256];
     const int k = blockIdx.x, t = threadIdx.x;
@@ -938,6 +953,11 @@ __global__ void __launch_bounds__(256) wide_flag_kernel(int D, int Dpad, int K, 
         const double a = 8.0 * est + eps * red[2][0] + 0.0625, w = eps * red[3][0];
         scra[k] = (float)fmin(isfinite(a) ? a : 1e30, 1e30);
         scrw[k] = (float)fmin(isfinite(w) ? w : 1e30, 1e30);
+        // with the leading product alone (the low halves of both operands dropped: 2^-11 of every term, twice)
+        const double eps_hi = 9.765625e-04;                  // 2^-10
+        const double ah = a + eps_hi * red[2][0], wh = w + eps_hi * red[3][0];
+        scra_hi[k] = (float)fmin(isfinite(ah) ? ah : 1e30, 1e30);
+        scrw_hi[k] = (float)fmin(isfinite(wh) ? wh : 1e30, 1e30);
     }
 }
 
@@ -1089,7 +1109,8 @@ __global__ void __launch_bounds__(256) wide_prepare_kernel(int D, int Dpad, int 
 __global__ void __launch_bounds__(1024) wide_cref_kernel(int rows, const int* __restrict__ flags, const float* __restrict__ tk,
                                                          const double* __restrict__ ckd, const int* __restrict__ comp_of,
                                                          const int* __restrict__ slot_of, const float* __restrict__ scra,
-                                                         const float* __restrict__ scrw, double* __restrict__ cref,
+                                                         const float* __restrict__ scrw, const float* __restrict__ scra_hi,
+                                                         const float* __restrict__ scrw_hi, int hi_mode, double* __restrict__ cref,
                                                          float2* __restrict__ tkck, float2* __restrict__ scr,
                                                          float* __restrict__ scr_e) {
     __shared__ double red[1024];
@@ -1105,14 +1126,19 @@ __global__ void __launch_bounds__(1024) wide_cref_kernel(int rows, const int* __
     }
     const double r = isfinite(red[0]) ? red[0] : 0.0;
     if (threadIdx.x == 0) *cref = r;
+    const int hi_start = ((((Kg + 255) & ~255) + flags[5]) + 255) & ~255;
     for (int k = threadIdx.x; k < rows; k += 1024) {
         const bool in = k < Kg && isfinite(ckd[k]);
         tkck[k] = make_float2(tk[k], in ? (float)(ckd[k] - r) : -CUDART_INF_F);
         const int c = comp_of[k];
         const bool listed = slot_of[k] >= 0 && c >= 0 && isfinite(ckd[k]);
-        scr[k] = listed ? make_float2((float)fmin(ckd[k] - r + (double)scra[c], 3e38), scrw[c])
+        // (hi_mode: the groups of 256 positions behind the first kind of listed components are screened by the leading
+        // product alone, with the allowances that go with it)
+        const bool hi = hi_mode != 0 && k >= hi_start;
+        const float ea = listed ? (hi ? scra_hi[c] : scra[c]) : 0.f, ew = listed ? (hi ? scrw_hi[c] : scrw[c]) : 0.f;
+        scr[k] = listed ? make_float2((float)fmin(ckd[k] - r + (double)ea, 3e38), ew)
                         : (in && c >= 0) ? make_float2(scra[c], scrw[c]) : make_float2(-CUDART_INF_F, 0.f);
-        scr_e[k] = listed ? scra[c] : 0.f;
+        scr_e[k] = ea;
     }
 }
 
@@ -1974,14 +2000,14 @@ WidePlan wide_plan(int D, int K, int num_sms) {
 }
 
 cudaError_t launch_prepare_wide(cudaStream_t s, int D, int K, const float* pi, const float* mu, const float* var,
-                                const WideBuffers& wb, float cond_limit, float min_weight) {
+                                const WideBuffers& wb, float cond_limit, float min_weight, bool hi_mode) {
     const WidePlan pl = wide_plan(D, K, 148);
     cudaError_t e = cudaMemsetAsync(wb.flags, 0, 8 * sizeof(int), s);
     if (e != cudaSuccess) return e;
     wide_scale_kernel<<<pl.Dpad, 128, 0, s>>>(D, K, pi, mu, var, wb.sd, wb.kap, wb.gd);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    wide_flag_kernel<<<K, 256, 0, s>>>(D, pl.Dpad, K, pi, mu, var, wb.sd, wb.kap, wb.gd, wb.illb, wb.scra, wb.scrw, cond_limit,
+    wide_flag_kernel<<<K, 256, 0, s>>>(D, pl.Dpad, K, pi, mu, var, wb.sd, wb.kap, wb.gd, wb.illb, wb.scra, wb.scrw, wb.scra_hi, wb.scrw_hi, cond_limit,
                                        min_weight, wb.flags);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
@@ -1993,7 +2019,7 @@ cudaError_t launch_prepare_wide(cudaStream_t s, int D, int K, const float* pi, c
         reinterpret_cast<__half*>(wb.p_lo), wb.tk, wb.ckd);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    wide_cref_kernel<<<1, 1024, 0, s>>>(pl.rows, wb.flags, wb.tk, wb.ckd, wb.comp_of, wb.slot_of, wb.scra, wb.scrw, wb.cref,
+    wide_cref_kernel<<<1, 1024, 0, s>>>(pl.rows, wb.flags, wb.tk, wb.ckd, wb.comp_of, wb.slot_of, wb.scra, wb.scrw, wb.scra_hi, wb.scrw_hi, hi_mode ? 1 : 0, wb.cref,
                                         reinterpret_cast<float2*>(wb.tkck), reinterpret_cast<float2*>(wb.scr), wb.scr_e);
     return cudaGetLastError();
 }
@@ -2100,7 +2126,7 @@ cudaError_t launch_transform_wide(cudaStream_t s, const float* X, int64_t n, int
 }
 
 cudaError_t launch_lse_wide(cudaStream_t s, int64_t n, int D, int K, int Kg, int n_listed, int n_slots, const WideBuffers& wb,
-                            int num_sms, int* status, int ntop) {
+                            int num_sms, int* status, int ntop, int hi_first_slots) {
     if (n < 1 || n > WIDE_PIECE || Kg < 0 || Kg > K || (Kg < 1 && n_listed < 1)) return cudaErrorInvalidValue;
     const WidePlan pl = wide_plan(D, K, num_sms);
     const int64_t rp = rows_padded_of(n);
@@ -2128,6 +2154,7 @@ cudaError_t launch_lse_wide(cudaStream_t s, int64_t n, int D, int K, int Kg, int
     p.scr = reinterpret_cast<const float2*>(wb.scr);
     p.scr_e = wb.scr_e; p.scr_mask = wb.scr_mask; p.slot_of = wb.slot_of; p.n2 = wb.n2; p.cand = wb.cand;
     p.cand_words = (n_slots + 31) / 32; p.scr_group = Kgp / 256; p.ctl = wb.ctl;
+    p.hi_group = (screen && hi_first_slots >= 0 && ntop == 2) ? (Kgp + hi_first_slots + 255) / 256 : 0x7fffffff;
     const int64_t ntiles = (n + WIDE_TILE - 1) / WIDE_TILE;
     const unsigned grid = (unsigned)(ntiles < num_sms ? ntiles : num_sms);
     if (ntop == 2) lse_wide_kernel<2><<<grid, WT_THREADS, L_SMEM, s>>>(p, tm_yhi, tm_ylo, tm_phi, tm_plo);

@@ -45,6 +45,8 @@ struct WideBuffers {
     float* illb;    // [Kpad] by component: > 0 for an ill-conditioned one
     float* scra;    // [Kpad] by component: bound of the error of its approximate log2 z at the centre ...
     float* scrw;    // [Kpad] ... and per unit of |x - g|^2
+    float* scra_hi; // [Kpad] the same two for the leading product alone (low halves of the operands dropped)
+    float* scrw_hi;
     int* flags;     // [8]: [0] any ill-conditioned component, [4] how many, [2] slots of the list, [5] slots of its first
                     //      kind, [6] evaluated components (positions [0, flags[6])); [1], [3], [7]: see launch_cand_count_wide
     int* ill_list;  // [WIDE_MAX_ILL] ascending indices of the ill-conditioned components
@@ -83,7 +85,9 @@ WidePlan wide_plan(int D, int K, int num_sms);
 // min_weight are flagged (flags[4] counts them), listed (flags[2], flags[5]) and placed behind the others (flags[6] =
 // how many the tensor passes evaluate); coefficient planes and constants by position.
 cudaError_t launch_prepare_wide(cudaStream_t s, int D, int K, const float* pi, const float* mu, const float* var,
-                                const WideBuffers& wb, float cond_limit, float min_weight);
+                                const WideBuffers& wb, float cond_limit, float min_weight, bool hi_mode = false);
+// hi_mode (only with every component listed): the groups of 256 positions behind the first kind of listed components get
+// the allowances of the leading product alone; launch_lse_wide must then be given hi_first_slots = flags[5].
 // n <= WIDE_PIECE points: X -> the fp16 planes of Y (rows up to the next multiple of 256 are written as zeros).
 cudaError_t launch_transform_wide(cudaStream_t s, const float* X, int64_t n, int D, const WideBuffers& wb, int* status);
 // The listed components' rows of the FP32 path's derived parameters packed into wb.mu_c / w2_c / c2d_c.
@@ -107,8 +111,10 @@ cudaError_t launch_cand_count_wide(cudaStream_t s, const WideBuffers& wb);
 // listed component whose approximate log2 z, raised by its error bound, comes within 2^-40 of the point's maximum, and
 // counts the marks in wb.ctl[0]; wb.n2, wb.cand (zeroed) and wb.ctl (zeroed) must have been prepared for the piece.
 // ntop (2, 6 or WIDE_MAX_TOP): how many of a point's largest approximate values go to wb.top.
+// hi_first_slots >= 0 (with parameters prepared in hi_mode): the slots of the list's first kind (flags[5]); the groups of
+// 256 positions behind them are screened by the leading product alone.
 cudaError_t launch_lse_wide(cudaStream_t s, int64_t n, int D, int K, int Kg, int n_listed, int n_slots, const WideBuffers& wb,
-                            int num_sms, int* status, int ntop = 2);
+                            int num_sms, int* status, int ntop = 2, int hi_first_slots = -1);
 // Top-m assignment of the n points of a piece from what launch_lse_wide (ntop >= m + 2; screened: it also marked the listed
 // pairs) and launch_norm_wide left in wb: idx [n][m], resp [n][m] (may be NULL); rows whose answer is not certain are appended to unc_rows
 // (unc_count += 1 each) and left unwritten.  mu, w2, c2d: the FP32 path's derived parameters.

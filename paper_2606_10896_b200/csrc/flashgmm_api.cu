@@ -34,7 +34,7 @@ struct ScratchLayout {
     size_t tc_phi, tc_plo, tc_tk, tc_ck, tc_sd, tc_kap, tc_gd, tc_illb, tc_flags, tc_xg, tc_xl, tc_partial, tc_llpart, tc_partial_bytes, tc_yhi, tc_ylo, tc_phirm, tc_plorm, tc_tkck, tc_illlist, tc_illcache, tc_decdim, tc_decw, tc_decmu;
     bool tc;
     // the tensor-core path for D > 128
-    size_t w_sd, w_kap, w_gd, w_phi, w_plo, w_tk, w_tkck, w_ckd, w_cref, w_illb, w_flags, w_yhi, w_ylo, w_logz, w_partial, w_llpart, w_illlist, w_muc, w_w2c, w_c2dc, w_statsc, w_top, w_logzx, w_compof, w_scra, w_scrw, w_scr, w_slotof, w_scrmask, w_n2, w_cand, w_candT, w_ctl, w_scre, w_slotcnt, w_heavyof, w_heavyslot, w_heavypart;
+    size_t w_sd, w_kap, w_gd, w_phi, w_plo, w_tk, w_tkck, w_ckd, w_cref, w_illb, w_flags, w_yhi, w_ylo, w_logz, w_partial, w_llpart, w_illlist, w_muc, w_w2c, w_c2dc, w_statsc, w_top, w_logzx, w_compof, w_scra, w_scrw, w_scr, w_slotof, w_scrmask, w_n2, w_cand, w_candT, w_ctl, w_scre, w_slotcnt, w_heavyof, w_heavyslot, w_heavypart, w_scrahi, w_scrwhi;
     size_t w_partial_bytes;
     bool wide;
 };
@@ -89,7 +89,7 @@ ScratchLayout scratch_layout(int D, int K, bool planes) {
         L.tc_ylo = take(TC_YPLANE_BYTES);
     }
     L.w_sd = L.w_kap = L.w_gd = L.w_phi = L.w_plo = L.w_tk = L.w_tkck = L.w_ckd = L.w_cref = L.w_illb = L.w_flags = L.w_yhi = L.w_ylo = L.w_logz = L.w_partial = L.w_llpart = L.w_illlist = L.w_muc = L.w_w2c = L.w_c2dc = L.w_statsc = L.w_top = L.w_logzx = 0;
-    L.w_compof = L.w_scra = L.w_scrw = L.w_scr = L.w_slotof = L.w_scrmask = L.w_n2 = L.w_cand = L.w_candT = L.w_ctl = L.w_scre = L.w_slotcnt = L.w_heavyof = L.w_heavyslot = L.w_heavypart = 0;
+    L.w_compof = L.w_scra = L.w_scrw = L.w_scr = L.w_slotof = L.w_scrmask = L.w_n2 = L.w_cand = L.w_candT = L.w_ctl = L.w_scre = L.w_slotcnt = L.w_heavyof = L.w_heavyslot = L.w_heavypart = L.w_scrahi = L.w_scrwhi = 0;
     L.w_partial_bytes = 0;
     L.wide = wide_supports(D, K) && planes;
     if (L.wide) {
@@ -117,6 +117,8 @@ ScratchLayout scratch_layout(int D, int K, bool planes) {
         L.w_candT = take(slots * WIDE_CANDT_WORDS * 4);
         L.w_ctl = take(32);
         L.w_scre = take((size_t)wp.rows * 4);
+        L.w_scrahi = take((size_t)wp.Kpad * 4);
+        L.w_scrwhi = take((size_t)wp.Kpad * 4);
         L.w_slotcnt = take(slots * 4);
         L.w_heavyof = take(slots * 4);
         L.w_heavyslot = take((size_t)WIDE_HEAVY_SLOTS * 4);
@@ -181,6 +183,7 @@ struct gmm_ctx {
     double wide_probe_limit = 0.0;   // automatic mode: "screen" while a sample of the points has at most this many marked pairs per
                                      // point (0: K D / 70000, or K D / 8192 below 128 points per component)
     bool wide_screen_all = false;    // the current step runs in "screen" mode
+    bool wide_hi = true;             // GMM_WIDE_HI=0: the screening mode forms all three products for every component
     int wide_sparse = 1;             // GMM_WIDE_SPARSE: 0 = the listed components always go through the dense FP32 kernels,
                                      // 1 = pair by pair unless sweep 1 marks too many pairs, 2 = always pair by pair (tests)
     int tc_n_ill = 0;                // ill-conditioned components at the last result that was read back (picks the filter)
@@ -274,6 +277,8 @@ struct gmm_ctx {
         b.candT = reinterpret_cast<unsigned*>(scratch + lay.w_candT);
         b.ctl = reinterpret_cast<int*>(scratch + lay.w_ctl);
         b.scr_e = reinterpret_cast<float*>(scratch + lay.w_scre);
+        b.scra_hi = reinterpret_cast<float*>(scratch + lay.w_scrahi);
+        b.scrw_hi = reinterpret_cast<float*>(scratch + lay.w_scrwhi);
         b.slot_cnt = reinterpret_cast<int*>(scratch + lay.w_slotcnt);
         b.heavy_of = reinterpret_cast<int*>(scratch + lay.w_heavyof);
         b.heavy_slot = reinterpret_cast<int*>(scratch + lay.w_heavyslot);
@@ -450,7 +455,7 @@ int prepare_and_choose(gmm_ctx* ctx, int64_t N, int D, int K, const float* pi, c
         // alternative (it would list most components as light) and the FP32 kernels cost K D / 2 ns per point: K D / 8192.
         const bool few_points = N < WIDE_AUTO_MIN_POINTS_PER_COMPONENT * K;
         if (ctx->wide_mode == 2 || (ctx->wide_mode == 0 && can_probe)) {
-            KL(launch_prepare_wide(ctx->stream, D, K, pi, mu, var, wb, limit, INFINITY));      // every component is listed
+            KL(launch_prepare_wide(ctx->stream, D, K, pi, mu, var, wb, limit, INFINITY, ctx->wide_hi));      // every component is listed
             ctx->launches += 4;
             CU(cudaMemcpyAsync(fl, wb.flags, sizeof(fl), cudaMemcpyDeviceToHost, ctx->stream));
             CU(cudaStreamSynchronize(ctx->stream));
@@ -463,7 +468,7 @@ int prepare_and_choose(gmm_ctx* ctx, int64_t N, int D, int K, const float* pi, c
                 CU(launch_cand_clear_wide(ctx->stream, np, n_list, wb));
                 KL(launch_norm_wide(ctx->stream, Xprobe, np, D, wb));
                 KL(launch_transform_wide(ctx->stream, Xprobe, np, D, wb, &ctx->result()->status));
-                KL(launch_lse_wide(ctx->stream, np, D, K, fl[6], fl[4], n_list, wb, ctx->sms, &ctx->result()->status));
+                KL(launch_lse_wide(ctx->stream, np, D, K, fl[6], fl[4], n_list, wb, ctx->sms, &ctx->result()->status, 2, ctx->wide_hi ? fl[5] : -1));
                 int marks = 0;
                 CU(cudaMemcpyAsync(&marks, wb.ctl, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
                 CU(cudaStreamSynchronize(ctx->stream));
@@ -568,7 +573,8 @@ int accumulate_points(gmm_ctx* ctx, int path, const float* X, int64_t n, int D, 
             }
             CHECK(prof_begin(ctx));
             KL(launch_transform_wide(ctx->stream, Xs, cnt, D, wb, &ctx->result()->status));
-            KL(launch_lse_wide(ctx->stream, cnt, D, K, Kg, screen ? n_listed : 0, n_ill, wb, ctx->sms, &ctx->result()->status));
+            KL(launch_lse_wide(ctx->stream, cnt, D, K, Kg, screen ? n_listed : 0, n_ill, wb, ctx->sms, &ctx->result()->status, 2,
+                               (all && ctx->wide_hi) ? ctx->wide_n_first : -1));
             if (ctx->wide_refine && !all) KL(launch_refine_wide(ctx->stream, Xs, cnt, D, K, mu, ctx->w2(), ctx->c2d(), wb));
             else CU(cudaMemcpyAsync(wb.logz_x, wb.logz, (size_t)cnt * 8, cudaMemcpyDeviceToDevice, ctx->stream));
             if (n_ill > 0) {
@@ -721,6 +727,7 @@ int gmm_create(gmm_ctx** out, int device, void* cuda_stream) {
     if (const char* e = std::getenv("GMM_WIDE_MIN_POINTS")) ctx->wide_min_points = std::atof(e);
     if (const char* e = std::getenv("GMM_WIDE_REFINE")) ctx->wide_refine = std::atoi(e) != 0;
     if (const char* e = std::getenv("GMM_WIDE_SPARSE")) ctx->wide_sparse = std::atoi(e);
+    if (const char* e = std::getenv("GMM_WIDE_HI")) ctx->wide_hi = std::atoi(e) != 0;
     if (const char* e = std::getenv("GMM_WIDE_MODE")) ctx->wide_mode = !std::strcmp(e, "sweeps") ? 1 : !std::strcmp(e, "screen") ? 2 : 0;
     if (const char* e = std::getenv("GMM_WIDE_PROBE_LIMIT")) ctx->wide_probe_limit = std::atof(e);
     if (const char* e = std::getenv("GMM_WIDE_PIECE")) {

@@ -80,7 +80,8 @@ struct LseParams {
     unsigned* cand;      // [n][cand_words]
     int cand_words;
     int scr_group;       // first group of 256 columns that holds listed components (they hold nothing else from there on)
-    int hi_group;        // from this group on only the leading product (Y_hi P_hi) is formed: screening with wider allowances
+    int hi_group;        // groups [hi_group, hi_end): only the leading product (Y_hi P_hi) is formed, with wider allowances
+    int hi_end;
     int* ctl;
 };
 
@@ -169,7 +170,7 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
             for (int g = 0; g < NG; ++g) {
                 const int nch = (NC - 2 * g < 2) ? (NC - 2 * g) : 2;
                 const bool screening = p.screen && g >= p.scr_group;
-                const bool hi_grp = g >= p.hi_group;          // (only screening groups are ever of this kind)
+                const bool hi_grp = g >= p.hi_group && g < p.hi_end;
                 if (screening) {
                     // What a pair is screened against: the point's maximum over the evaluated components (final by now; the
                     // two warpgroups merge theirs at the first screening group) and the largest LOWER bound among the listed
@@ -238,8 +239,8 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
 #pragma unroll
                             for (int j = 0; j < 32; j += 2) {
                                 const float4 q = __ldg(tc4 + (j >> 1));          // (t, c) of two components; same address in every lane
-                                l[j] = fmaf(__uint_as_float(v[j]) + __uint_as_float(vc[j]), q.x, q.y);
-                                l[j + 1] = fmaf(__uint_as_float(v[j + 1]) + __uint_as_float(vc[j + 1]), q.z, q.w);
+                                l[j] = fmaf(hi_grp ? __uint_as_float(v[j]) : __uint_as_float(v[j]) + __uint_as_float(vc[j]), q.x, q.y);
+                                l[j + 1] = fmaf(hi_grp ? __uint_as_float(v[j + 1]) : __uint_as_float(v[j + 1]) + __uint_as_float(vc[j + 1]), q.z, q.w);
                                 bmax = fmaxf(bmax, fmaxf(l[j], l[j + 1]));
                             }
                             if (bmax > m_run) {
@@ -346,7 +347,7 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
             for (int gq = 0; gq < NG && ok; ++gq) {
                 const int nch = (NC - 2 * gq < 2) ? (NC - 2 * gq) : 2;
                 for (int z = 0; z < NZ && ok; ++z) {
-                    const bool hi_only = gq >= p.hi_group;
+                    const bool hi_only = gq >= p.hi_group && gq < p.hi_end;
                     ok = item(&tm_yhi, &tm_ylo, row0, z, false, hi_only);
                     for (int c = 0; c < nch && ok; ++c) ok = item(&tm_phi, &tm_plo, (2 * gq + c) * 128, z, true, hi_only);
                 }
@@ -391,7 +392,7 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
                             const uint32_t d = tmem + c * 128, dc = tmem + 256 + c * 128;
                             // the two small cross products into their own accumulator, the leading product into the main one:
                             // the same three chains, in the same order, as the E-step of sweep 2
-                            if (gq < p.hi_group) {
+                            if (!(gq >= p.hi_group && gq < p.hi_end)) {
 #pragma unroll
                                 for (int j = 0; j < 4; ++j) mma_ss(dc, ah + ((j * 32) >> 4), bl + ((j * 32) >> 4), idesc, (z > 0 || j > 0) ? 1u : 0u);
 #pragma unroll
@@ -1134,10 +1135,11 @@ __global__ void __launch_bounds__(1024) wide_cref_kernel(int rows, const int* __
         const bool listed = slot_of[k] >= 0 && c >= 0 && isfinite(ckd[k]);
         // (hi_mode: the groups of 256 positions behind the first kind of listed components are screened by the leading
         // product alone, with the allowances that go with it)
-        const bool hi = hi_mode != 0 && k >= hi_start;
+        const bool hi = hi_mode == 1 && k >= hi_start;
         const float ea = listed ? (hi ? scra_hi[c] : scra[c]) : 0.f, ew = listed ? (hi ? scrw_hi[c] : scrw[c]) : 0.f;
         scr[k] = listed ? make_float2((float)fmin(ckd[k] - r + (double)ea, 3e38), ew)
-                        : (in && c >= 0) ? make_float2(scra[c], scrw[c]) : make_float2(-CUDART_INF_F, 0.f);
+                        : (in && c >= 0) ? (hi_mode == 2 ? make_float2(scra_hi[c], scrw_hi[c]) : make_float2(scra[c], scrw[c]))
+                                         : make_float2(-CUDART_INF_F, 0.f);
         scr_e[k] = ea;
     }
 }
@@ -2000,7 +2002,7 @@ WidePlan wide_plan(int D, int K, int num_sms) {
 }
 
 cudaError_t launch_prepare_wide(cudaStream_t s, int D, int K, const float* pi, const float* mu, const float* var,
-                                const WideBuffers& wb, float cond_limit, float min_weight, bool hi_mode) {
+                                const WideBuffers& wb, float cond_limit, float min_weight, int hi_mode) {
     const WidePlan pl = wide_plan(D, K, 148);
     cudaError_t e = cudaMemsetAsync(wb.flags, 0, 8 * sizeof(int), s);
     if (e != cudaSuccess) return e;
@@ -2019,7 +2021,7 @@ cudaError_t launch_prepare_wide(cudaStream_t s, int D, int K, const float* pi, c
         reinterpret_cast<__half*>(wb.p_lo), wb.tk, wb.ckd);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    wide_cref_kernel<<<1, 1024, 0, s>>>(pl.rows, wb.flags, wb.tk, wb.ckd, wb.comp_of, wb.slot_of, wb.scra, wb.scrw, wb.scra_hi, wb.scrw_hi, hi_mode ? 1 : 0, wb.cref,
+    wide_cref_kernel<<<1, 1024, 0, s>>>(pl.rows, wb.flags, wb.tk, wb.ckd, wb.comp_of, wb.slot_of, wb.scra, wb.scrw, wb.scra_hi, wb.scrw_hi, hi_mode, wb.cref,
                                         reinterpret_cast<float2*>(wb.tkck), reinterpret_cast<float2*>(wb.scr), wb.scr_e);
     return cudaGetLastError();
 }
@@ -2099,11 +2101,11 @@ cudaError_t launch_cand_mstep_wide(cudaStream_t s, const float* X, int64_t n, in
 
 cudaError_t launch_assign_refine_wide(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu, const float* w2,
                                       const double* c2d, int n_slots, bool screened, const WideBuffers& wb, int ntop, int m,
-                                      int32_t* idx, float* resp, int32_t* unc_rows, int* unc_count, bool index_only) {
+                                      int32_t* idx, float* resp, int32_t* unc_rows, int* unc_count, bool index_only, bool hi) {
     if (m < 1 || m > GMM_MAX_TOPM || m > ntop) return cudaErrorInvalidValue;
     WideAssignArgs g;
     g.X = X; g.n = n; g.D = D; g.K = K; g.mu = mu; g.w2 = w2; g.c2d = c2d;
-    g.comp_of = wb.comp_of; g.top = wb.top; g.logz = wb.logz; g.cref = wb.cref; g.n2 = wb.n2; g.scra = wb.scra; g.scrw = wb.scrw;
+    g.comp_of = wb.comp_of; g.top = wb.top; g.logz = wb.logz; g.cref = wb.cref; g.n2 = wb.n2; g.scra = hi ? wb.scra_hi : wb.scra; g.scrw = hi ? wb.scrw_hi : wb.scrw;
     g.cand = screened ? wb.cand : nullptr; g.cand_words = (n_slots + 31) / 32; g.list = wb.ill_list;
     g.mu_c = wb.mu_c; g.w2_c = wb.w2_c; g.c2d_c = wb.c2d_c; g.ctl = screened ? wb.ctl : nullptr;
     g.m = m; g.idx = idx; g.resp = resp; g.unc_rows = unc_rows; g.unc_count = unc_count; g.index_only = index_only;
@@ -2154,7 +2156,9 @@ cudaError_t launch_lse_wide(cudaStream_t s, int64_t n, int D, int K, int Kg, int
     p.scr = reinterpret_cast<const float2*>(wb.scr);
     p.scr_e = wb.scr_e; p.scr_mask = wb.scr_mask; p.slot_of = wb.slot_of; p.n2 = wb.n2; p.cand = wb.cand;
     p.cand_words = (n_slots + 31) / 32; p.scr_group = Kgp / 256; p.ctl = wb.ctl;
-    p.hi_group = (screen && hi_first_slots >= 0 && ntop == 2) ? (Kgp + hi_first_slots + 255) / 256 : 0x7fffffff;
+    p.hi_group = 0x7fffffff; p.hi_end = 0x7fffffff;
+    if (ntop == 2 && screen && hi_first_slots >= 0) p.hi_group = (Kgp + hi_first_slots + 255) / 256;        // the EM step's screening mode
+    if (ntop != 2 && hi_first_slots >= 0) { p.hi_group = 0; p.hi_end = Kgp / 256; }                         // the assignment's evaluated groups
     const int64_t ntiles = (n + WIDE_TILE - 1) / WIDE_TILE;
     const unsigned grid = (unsigned)(ntiles < num_sms ? ntiles : num_sms);
     if (ntop == 2) lse_wide_kernel<2><<<grid, WT_THREADS, L_SMEM, s>>>(p, tm_yhi, tm_ylo, tm_phi, tm_plo);

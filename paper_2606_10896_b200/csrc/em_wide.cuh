@@ -85,9 +85,11 @@ WidePlan wide_plan(int D, int K, int num_sms);
 // min_weight are flagged (flags[4] counts them), listed (flags[2], flags[5]) and placed behind the others (flags[6] =
 // how many the tensor passes evaluate); coefficient planes and constants by position.
 cudaError_t launch_prepare_wide(cudaStream_t s, int D, int K, const float* pi, const float* mu, const float* var,
-                                const WideBuffers& wb, float cond_limit, float min_weight, bool hi_mode = false);
-// hi_mode (only with every component listed): the groups of 256 positions behind the first kind of listed components get
-// the allowances of the leading product alone; launch_lse_wide must then be given hi_first_slots = flags[5].
+                                const WideBuffers& wb, float cond_limit, float min_weight, int hi_mode = 0);
+// hi_mode 1 (only with every component listed): the groups of 256 positions behind the first kind of listed components
+// get the allowances of the leading product alone; launch_lse_wide must then be given hi_first_slots = flags[5].
+// hi_mode 2 (the assignment): the evaluated components get them; launch_lse_wide (ntop > 2) is given hi_first_slots = 0
+// and launch_assign_refine_wide hi = true.
 // n <= WIDE_PIECE points: X -> the fp16 planes of Y (rows up to the next multiple of 256 are written as zeros).
 cudaError_t launch_transform_wide(cudaStream_t s, const float* X, int64_t n, int D, const WideBuffers& wb, int* status);
 // The listed components' rows of the FP32 path's derived parameters packed into wb.mu_c / w2_c / c2d_c.
@@ -120,7 +122,8 @@ cudaError_t launch_lse_wide(cudaStream_t s, int64_t n, int D, int K, int Kg, int
 // (unc_count += 1 each) and left unwritten.  mu, w2, c2d: the FP32 path's derived parameters.
 cudaError_t launch_assign_refine_wide(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu, const float* w2,
                                       const double* c2d, int n_slots, bool screened, const WideBuffers& wb, int ntop, int m,
-                                      int32_t* idx, float* resp, int32_t* unc_rows, int* unc_count, bool index_only);
+                                      int32_t* idx, float* resp, int32_t* unc_rows, int* unc_count, bool index_only,
+                                      bool hi = false);
 // wb.n2[i] = |x_i - g|^2 for the n points of a piece.
 cudaError_t launch_norm_wide(cudaStream_t s, const float* X, int64_t n, int D, const WideBuffers& wb);
 // Clears wb.ctl, the n rows of wb.cand and the n_slots rows of wb.candT before a piece's first sweep.

@@ -455,7 +455,7 @@ int prepare_and_choose(gmm_ctx* ctx, int64_t N, int D, int K, const float* pi, c
         // alternative (it would list most components as light) and the FP32 kernels cost K D / 2 ns per point: K D / 8192.
         const bool few_points = N < WIDE_AUTO_MIN_POINTS_PER_COMPONENT * K;
         if (ctx->wide_mode == 2 || (ctx->wide_mode == 0 && can_probe)) {
-            KL(launch_prepare_wide(ctx->stream, D, K, pi, mu, var, wb, limit, INFINITY, ctx->wide_hi));      // every component is listed
+            KL(launch_prepare_wide(ctx->stream, D, K, pi, mu, var, wb, limit, INFINITY, ctx->wide_hi ? 1 : 0));      // every component is listed
             ctx->launches += 4;
             CU(cudaMemcpyAsync(fl, wb.flags, sizeof(fl), cudaMemcpyDeviceToHost, ctx->stream));
             CU(cudaStreamSynchronize(ctx->stream));
@@ -1039,7 +1039,11 @@ int assign_topm_impl(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, cons
         if (want) {
             const WideBuffers wb = ctx->wide();
             const float limit = ctx->tc_cond_limit >= 0.f ? ctx->tc_cond_limit : 0.01f;
-            KL(launch_prepare_wide(ctx->stream, D, K, pi, mu, var, wb, limit, 0.f));
+            // (indices only: the sweep forms the leading fp16 product alone for the evaluated components - a third of the tensor
+            // work - and ranks by correspondingly wider bounds; with responsibilities asked for, the approximate log Z has to
+            // be good and all three products are formed)
+            const bool hi = index_only && ctx->wide_hi;
+            KL(launch_prepare_wide(ctx->stream, D, K, pi, mu, var, wb, limit, 0.f, hi ? 2 : 0));
             ctx->launches += 4;
             int fl[8];
             CU(cudaMemcpyAsync(fl, wb.flags, sizeof(fl), cudaMemcpyDeviceToHost, ctx->stream));
@@ -1069,10 +1073,10 @@ int assign_topm_impl(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, cons
                     CHECK(prof_begin(ctx));
                     KL(launch_norm_wide(ctx->stream, Xs, cnt, D, wb));
                     KL(launch_transform_wide(ctx->stream, Xs, cnt, D, wb, &ctx->result()->status));
-                    KL(launch_lse_wide(ctx->stream, cnt, D, K, Kg, screen ? n_ill : 0, n_list, wb, ctx->sms, &ctx->result()->status, ntop));
+                    KL(launch_lse_wide(ctx->stream, cnt, D, K, Kg, screen ? n_ill : 0, n_list, wb, ctx->sms, &ctx->result()->status, ntop, hi ? 0 : -1));
                     if (screen) KL(launch_cand_gate_wide(ctx->stream, wb, ctx->wide_sparse >= 2 ? ((long long)1 << 62) : (long long)cnt * n_list / 64));
                     KL(launch_assign_refine_wide(ctx->stream, Xs, cnt, D, K, mu, ctx->w2(), ctx->c2d(), n_list, screen, wb, ntop, m, idx_p, resp_p,
-                                                 unc_rows, unc_count, index_only));
+                                                 unc_rows, unc_count, index_only, hi));
                     // the rows left uncertain, against all K components; and the whole piece if its marked pairs were too many
                     KL(launch_topm_fp32(ctx->stream, Xs, cnt, D, K, mu, ctx->w2(), ctx->c2d(), ctx->center(), m, idx_p, resp_p, nullptr, unc_rows, unc_count));
                     if (screen) KL(launch_topm_fp32(ctx->stream, Xs, cnt, D, K, mu, ctx->w2(), ctx->c2d(), ctx->center(), m, idx_p, resp_p, wb.ctl + 1));

@@ -262,6 +262,10 @@ def main():
             timed_counts = exact_counts[-args.steps:]
             kg_share = 1.0 - (sum(timed_counts) / len(timed_counts) / K if timed_counts else 0.0)
             executed_factor = (12.0 + 24.0 * kg_share) / 8.0
+            if kg_share <= 0.01:
+                # screening mode: the sweep forms three products for the narrow components and one for the others (how many of
+                # each is not reported), and the statistics come from exact fp32 evaluations: no executed-work figure
+                executed_factor = None
             timed_launch = ("per piece of 2^17 points: wide_transform_kernel + lse_wide_kernel (+ em_wide_kernel in the two-sweep mode), plus the exact "
                             "evaluation of the components left out of the tensor passes (all inside the timed bracket)")
             traffic_key = "wide" if kg_share > 0.01 else "wide_screen"     # (no component in the second sweep: the screening mode)
@@ -297,7 +301,7 @@ def main():
         "traffic": traffic, "traffic_source": traffic_source, "peak_source": peak_note, "kernel_ms_per_step": kern_ms_step,
         "kernel_launches_per_step": kern_n / args.steps, "timed_launch": timed_launch,
         "algorithmic_flop_per_step": flops_step,
-        "frac_executed": achieved_tf * executed_factor / peak_tf,
+        "frac_executed": (achieved_tf * executed_factor / peak_tf) if executed_factor else None,
         "frac_fp32_accurate_tensor": (achieved_tf / (peak_tf / 3.0)) if bound == "tensor" else None,
         "hbm_frac": (bytes_X + 2 * K * D * 4) / (kern_ms_step * 1e-3) / 1e9 / peaks["hbm_gbs"],
         "ex2_per_s": N * K * ((1.0 + kg_share) if (wide and path_used == fg.GMM_PATH_TENSOR) else 1) / (kern_ms_step * 1e-3),

@@ -38,6 +38,7 @@
 #include <cuda.h>
 #include <cuda_fp16.h>
 #include <math_constants.h>
+#include <cstdlib>
 
 #define TC_WAIT_LIMIT_NS 2000000000ull
 #include "tc_prims.cuh"
@@ -53,11 +54,21 @@ constexpr float RSCALE = TC_RSCALE;
 
 // ------------------------------------------------------------------------------------------------------------------
 // Sweep 1
-constexpr int L_SLOTS = 6;                          // two steps (Y atom + two coefficient atoms) in flight
-constexpr int L_BAR = L_SLOTS * SLOT;
+// The ring holds four stages of 48 KB: one plane's atoms of a contraction step, [Y atom | coefficient atoms of the group's
+// two chunks] (the two chunks adjacent: one operand of 256 rows).  A step of a group that forms all three products takes
+// two stages (hi planes, lo planes), a step of a leading-product group one.  One barrier pair and one commit per stage:
+// with a barrier pair per atom the two single-lane loops (loads, MMAs) took 2000 cycles per step of 516 cycles of MMAs.
+constexpr int HSLOT = 16384;
+constexpr int L_STAGE = 3 * HSLOT;
+constexpr int L_SLOTS = 4;
+constexpr int L_BAR = L_SLOTS * L_STAGE;
 constexpr int L_MERGE = L_BAR + 256;                // 128 x 8 bytes: (max, sum) pairs of warpgroup 1, later the log-likelihood terms
 constexpr int L_SMEM = L_MERGE + 1024 + 1024;
-enum { LB_FULL = 0, LB_EMPTY = L_SLOTS, LB_LFULL = 2 * L_SLOTS, LB_LEMPTY, LB_FINAL, LB_COUNT };
+// LB_LFULL, LB_LEMPTY: one pair per half of the accumulator columns.  A group that forms all three products fills both
+// halves (main products in [0, 256), cross products in [256, 512)); a leading-product group fills one, so that the next
+// group's products run while the softmax warps read this one's.
+enum { LB_FULL = 0, LB_EMPTY = L_SLOTS, LB_LFULL = 2 * L_SLOTS, LB_LEMPTY = 2 * L_SLOTS + 2, LB_FINAL = 2 * L_SLOTS + 4, LB_COUNT };
+static_assert(LB_COUNT * 8 <= 256, "barriers");
 
 struct LseParams {
     int64_t n;
@@ -82,6 +93,7 @@ struct LseParams {
     int scr_group;       // first group of 256 columns that holds listed components (they hold nothing else from there on)
     int hi_group;        // groups [hi_group, hi_end): only the leading product (Y_hi P_hi) is formed, with wider allowances
     int hi_end;
+    int pre_pass;        // 1: before a tile's sweep proper, the groups from hi_group on are swept once for their lower bounds only
     int* ctl;
 };
 
@@ -122,12 +134,25 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
     double* ll_s = reinterpret_cast<double*>(smem + L_MERGE);      // after the last tile
     __shared__ float top_s[128][2 * NTOP + 1];
     __shared__ float xm_s[256];
+    // Per-component constants of the group at hand, one copy per warpgroup and two buffers (a warpgroup fills one while its
+    // slower warps may still read the other): (t, c, screening offset, screening slope), the allowance alone, the chunk masks.
+    // Read from global memory inside the loops over the accumulators they cost a trip to L2 per pair of components (the
+    // shared-memory ring leaves almost no L1).
+    __shared__ float4 tab_s[2][2][128];
+    __shared__ float tabe_s[2][2][128];
+    __shared__ int tabm_s[2][2][4];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int64_t ntiles = (p.n + WIDE_TILE - 1) / WIDE_TILE;
     const int64_t ntl = ((int64_t)blockIdx.x < ntiles) ? (ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
     const int NC = p.NC, NZ = p.NZ;
     const int NG = (NC + 1) >> 1;                        // groups of two chunks
+    // A tile's steps, the same for every role: with pre_pass the groups from hi_group on once for their lower bounds (so that
+    // the threshold is final before anything is marked), then every group.
+    const int npre = (p.pre_pass && p.hi_group < NG) ? NG - p.hi_group : 0;
+    const int nsteps = npre + NG;
+    auto step_group = [&](int t) { return t < npre ? p.hi_group + t : t - npre; };
+    auto leading_only = [&](int g) { return g >= p.hi_group && g < p.hi_end; };
 
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L_BAR);
     auto BAR = [&](int i) { return smem_u32(&bars[i]); };
@@ -135,8 +160,7 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
         abort_s = 0;
         drain_s = 0;
         for (int s = 0; s < L_SLOTS; ++s) { bar_init(BAR(LB_FULL + s), 1); bar_init(BAR(LB_EMPTY + s), 1); }
-        bar_init(BAR(LB_LFULL), 1);
-        bar_init(BAR(LB_LEMPTY), 256);
+        for (int b = 0; b < 2; ++b) { bar_init(BAR(LB_LFULL + b), 1); bar_init(BAR(LB_LEMPTY + b), 256); }
         bar_init(BAR(LB_FINAL), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -157,8 +181,28 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
         const uint32_t lane_addr = ((uint32_t)(wq * 32)) << 16;
         const int pt = wq * 32 + lane;                       // point within the tile
         const double cref = *p.cref;
-        uint32_t uses = 0;
+        uint32_t ub0 = 0, ub1 = 0, tcount = 0;               // uses of the two accumulator halves; tables staged so far
+        int nb = 0;                                          // the half the next leading-product group takes
         double ll_acc = 0.0;
+        float2 n_tk = make_float2(0.f, 0.f), n_sc = make_float2(0.f, 0.f);
+        float n_se = 0.f;
+        int n_mask = 0;
+        auto table_load = [&](int g) {                       // this thread's component of the warpgroup's chunk of group g
+            if (2 * g + grp < NC) {
+                const int col = (2 * g + grp) * 128 + pt;
+                n_tk = __ldg(p.tkck + col);
+                if (p.screen || NTOP > 2) n_sc = __ldg(p.scr + col);
+                if (p.screen) {
+                    n_se = __ldg(p.scr_e + col);
+                    if (pt < 4) n_mask = __ldg(p.scr_mask + (col >> 5) + pt);
+                }
+            }
+        };
+        auto table_store = [&](int tb) {
+            tab_s[tb][grp][pt] = make_float4(n_tk.x, n_tk.y, n_sc.x, n_sc.y);
+            tabe_s[tb][grp][pt] = n_se;
+            if (pt < 4) tabm_s[tb][grp][pt] = n_mask;
+        };
         for (int64_t i = 0; i < ntl; ++i) {
             const int64_t row = (blockIdx.x + i * gridDim.x) * WIDE_TILE + pt;
             float m_run = -1e30f, s_run = 0.f;               // finite start: blocks of -inf logits must not make NaN
@@ -167,19 +211,33 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
             int nhit = 0;
             WideTop<NTOP> tl;                                // the largest logits of this thread's chunks, and where
             tl.init();
-            for (int g = 0; g < NG; ++g) {
+            table_load(step_group(0));
+            table_store((int)(tcount & 1u));
+            for (int t = 0; t < nsteps; ++t) {
+                const int ph = t < npre ? 0 : 1;             // 0: lower bounds only
+                const int g = step_group(t);
                 const int nch = (NC - 2 * g < 2) ? (NC - 2 * g) : 2;
                 const bool screening = p.screen && g >= p.scr_group;
-                const bool hi_grp = g >= p.hi_group && g < p.hi_end;
+                const bool hi_grp = leading_only(g);
+                const int tb = (int)(tcount & 1u);
+                ++tcount;
+                named_bar_sync(4 + grp, 128);                // the group's table is in place (and the other buffer free)
+                const float4* tab = tab_s[tb][grp];
+                if (t == 0 && npre > 0) {                    // the tile's first use of the exchange slots
+                    xm_s[grp * 128 + pt] = thr_base;
+                    named_bar_sync(3, 256);
+                }
                 if (screening) {
                     // What a pair is screened against: the point's maximum over the evaluated components (final by now; the
                     // two warpgroups merge theirs at the first screening group) and the largest LOWER bound among the listed
                     // components seen so far (each warpgroup publishes its own after every group and picks up the other's:
                     // a value that is a little old is still a valid bound).
-                    if (g == p.scr_group) {
-                        xm_s[grp * 128 + pt] = m_run;
+                    if (ph == 1 && g == p.scr_group) {
+                        const float mine = fmaxf(m_run, thr_base);
+                        named_bar_sync(3, 256);               // (nobody still reads the slots of an earlier phase)
+                        xm_s[grp * 128 + pt] = mine;
                         named_bar_sync(3, 256);
-                        thr_base = fmaxf(m_run, xm_s[(grp ^ 1) * 128 + pt]);
+                        thr_base = fmaxf(mine, xm_s[(grp ^ 1) * 128 + pt]);
                         named_bar_sync(3, 256);
                         xm_s[grp * 128 + pt] = thr_base;
                     } else {
@@ -187,10 +245,23 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
                         thr_base = fmaxf(thr_base, xm_s[(grp ^ 1) * 128 + pt]);
                     }
                 }
-                const bool got = bar_wait(BAR(LB_LFULL), uses & 1u, abort_flag, p.status, false);
+                int half = 0;
+                bool got;
+                if (hi_grp) {
+                    half = nb;
+                    nb ^= 1;
+                    got = bar_wait(BAR(LB_LFULL + half), (half ? ub1 : ub0) & 1u, abort_flag, p.status, false);
+                    if (half) ++ub1; else ++ub0;
+                } else {
+                    got = bar_wait(BAR(LB_LFULL), ub0 & 1u, abort_flag, p.status, false);
+                    got = bar_wait(BAR(LB_LFULL + 1), ub1 & 1u, abort_flag, p.status, false) && got;
+                    ++ub0;
+                    ++ub1;
+                }
                 const bool ok = __all_sync(0xffffffffu, got);
                 fence_after();
-                ++uses;
+                if (t + 1 < nsteps) table_load(step_group(t + 1));    // (in flight during this group's pass)
+                const uint32_t acc = tmem + (uint32_t)(half * 256);
                 if (ok) {
                     {
                         const int c = grp;
@@ -198,23 +269,23 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
 #pragma unroll 1
                         for (int sub = 0; sub < 4; ++sub) {
                             uint32_t v[32], vc[32];
-                            tmem_ld32(tmem + c * 128 + sub * 32 + lane_addr, v);
-                            tmem_ld32(tmem + 256 + c * 128 + sub * 32 + lane_addr, vc);
+                            tmem_ld32(acc + c * 128 + sub * 32 + lane_addr, v);
+                            if (!hi_grp) tmem_ld32(tmem + 256 + c * 128 + sub * 32 + lane_addr, vc);
                             tmem_wait_ld();
                             const int col0 = (2 * g + c) * 128 + sub * 32;
-                            const float4* tc4 = reinterpret_cast<const float4*>(p.tkck + col0);
+                            const float4* tb4 = tab + sub * 32;
                             if (screening) {
                                 // Columns of listed components (they take no part in the sums): their approximate values,
                                 // raised by what they can be wrong by, tell which pairs can matter at all.  The point's
                                 // maximum over the evaluated components is final by now.  (!(a < b): a NaN passes.)
-                                if (__ldg(p.scr_mask + (col0 >> 5)) != 0 && row < p.n) {
-                                    const float4* sc4 = reinterpret_cast<const float4*>(p.scr + col0);
-                                    const float2* se2 = reinterpret_cast<const float2*>(p.scr_e + col0);
+                                if (tabm_s[tb][grp][sub] != 0 && row < p.n) {
+                                    const float2* se2 = reinterpret_cast<const float2*>(&tabe_s[tb][grp][sub * 32]);
 #pragma unroll
                                     for (int j = 0; j < 32; j += 2) {
-                                        const float4 q = __ldg(tc4 + (j >> 1));
-                                        const float4 sq = __ldg(sc4 + (j >> 1));
-                                        const float2 se = __ldg(se2 + (j >> 1));
+                                        const float4 t0 = tb4[j], t1 = tb4[j + 1];
+                                        const float4 q = make_float4(t0.x, t0.y, t1.x, t1.y);
+                                        const float4 sq = make_float4(t0.z, t0.w, t1.z, t1.w);
+                                        const float2 se = se2[j >> 1];
                                         const float a0 = hi_grp ? __uint_as_float(v[j]) : __uint_as_float(v[j]) + __uint_as_float(vc[j]);
                                         const float a1 = hi_grp ? __uint_as_float(v[j + 1]) : __uint_as_float(v[j + 1]) + __uint_as_float(vc[j + 1]);
                                         const float u0 = fmaf(a0, q.x, fmaf(sq.y, nrm, sq.x));
@@ -222,6 +293,7 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
                                         // lower bounds: the upper bound minus twice the allowance (fmaxf drops a NaN)
                                         thr_base = fmaxf(thr_base, fmaxf(u0 - 2.f * fmaf(sq.y, nrm, se.x), u1 - 2.f * fmaf(sq.w, nrm, se.y)));
                                         const float thr = thr_base - 40.f;
+                                        if (ph == 0) continue;                          // (lower bounds only)
                                         if (!(u0 < thr) && sq.x > -CUDART_INF_F) {
                                             const int sl = __ldg(p.slot_of + col0 + j);
                                             if (sl >= 0) { atomicOr(p.cand + row * p.cand_words + (sl >> 5), 1u << (sl & 31)); ++nhit; }
@@ -238,7 +310,8 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
                             float bmax = -CUDART_INF_F;
 #pragma unroll
                             for (int j = 0; j < 32; j += 2) {
-                                const float4 q = __ldg(tc4 + (j >> 1));          // (t, c) of two components; same address in every lane
+                                const float4 t0 = tb4[j], t1 = tb4[j + 1];       // same address in every lane
+                                const float4 q = make_float4(t0.x, t0.y, t1.x, t1.y);
                                 l[j] = fmaf(hi_grp ? __uint_as_float(v[j]) : __uint_as_float(v[j]) + __uint_as_float(vc[j]), q.x, q.y);
                                 l[j + 1] = fmaf(hi_grp ? __uint_as_float(v[j + 1]) : __uint_as_float(v[j + 1]) + __uint_as_float(vc[j + 1]), q.z, q.w);
                                 bmax = fmaxf(bmax, fmaxf(l[j], l[j + 1]));
@@ -255,17 +328,18 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
                             } else {
                                 // the assignment ranks by an UPPER bound of the exact value (approximate value + what it can be
                                 // wrong by for this point): what is not reported then lies below the last reported bound
-                                const float4* sc4 = reinterpret_cast<const float4*>(p.scr + col0);
                                 float bub = -CUDART_INF_F;
 #pragma unroll
                                 for (int j = 0; j < 32; j += 2) {
-                                    const float4 sq = __ldg(sc4 + (j >> 1));
+                                    const float4 t0 = tb4[j], t1 = tb4[j + 1];
+                                    const float4 sq = make_float4(t0.z, t0.w, t1.z, t1.w);
                                     bub = fmaxf(bub, fmaxf(l[j] + fmaf(sq.y, nrm, sq.x), l[j + 1] + fmaf(sq.w, nrm, sq.z)));
                                 }
                                 if (bub > tl.a[NTOP - 1]) {
 #pragma unroll
                                     for (int j = 0; j < 32; j += 2) {
-                                        const float4 sq = __ldg(sc4 + (j >> 1));
+                                        const float4 t0 = tb4[j], t1 = tb4[j + 1];
+                                        const float4 sq = make_float4(t0.z, t0.w, t1.z, t1.w);
                                         tl.insert(l[j] + fmaf(sq.y, nrm, sq.x), col0 + j);
                                         tl.insert(l[j + 1] + fmaf(sq.w, nrm, sq.z), col0 + j + 1);
                                     }
@@ -283,7 +357,9 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
                     }
                 }
                 fence_before();
-                bar_arrive(BAR(LB_LEMPTY));
+                if (hi_grp) bar_arrive(BAR(LB_LEMPTY + half));
+                else { bar_arrive(BAR(LB_LEMPTY)); bar_arrive(BAR(LB_LEMPTY + 1)); }
+                if (t + 1 < nsteps) table_store((int)(tcount & 1u));
             }
             // merge the two warpgroups' pairs; warpgroup 0 writes log2 Z and the two leading candidates
             if (grp == 1) {
@@ -319,11 +395,12 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
         }
     } else if (warp == WT_PRODUCER) {
         // =========================== producer warp (TMA) ===========================
-        // Item order = order of use: per (tile, group, atom z) the tile's Y atom, then the group's coefficient atoms.
+        // Stage order = order of use: per (tile, step of the tile, atom z) the hi planes' stage, then (unless the group forms
+        // the leading product only) the lo planes' stage.
         int64_t g = 0;
         bool ok = true;
         const uint64_t pol_keep = l2_policy_evict_last(), pol_stream = l2_policy_evict_first();
-        auto item = [&](const CUtensorMap* mh, const CUtensorMap* ml, int32_t row, int32_t z, bool keep, bool hi_only) -> bool {
+        auto stage = [&](const CUtensorMap* my, const CUtensorMap* mp, int32_t yrow, int32_t prow, int nch, int32_t z) -> bool {
             const int slot = (int)(g % L_SLOTS);
             const int64_t use = g / L_SLOTS;
             if (use > 0) {
@@ -332,11 +409,12 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
                 if (!__shfl_sync(0xffffffffu, w, 0)) return false;
             }
             if (elect_one()) {
-                const uint32_t dst = smem_u32(smem + slot * SLOT);
-                bar_expect_tx(BAR(LB_FULL + slot), hi_only ? SLOT / 2 : SLOT);
-                // the coefficient atoms are read by every CTA for every tile, the tile's own atoms once
-                tma_load_3d_hint(dst, mh, 0, row, z, BAR(LB_FULL + slot), keep ? pol_keep : pol_stream);
-                if (!hi_only) tma_load_3d_hint(dst + SLOT / 2, ml, 0, row, z, BAR(LB_FULL + slot), keep ? pol_keep : pol_stream);
+                const uint32_t dst = smem_u32(smem + slot * L_STAGE);
+                bar_expect_tx(BAR(LB_FULL + slot), (uint32_t)((1 + nch) * HSLOT));
+                // the coefficient atoms are read by every CTA for every tile, the tile's own atoms once per group
+                tma_load_3d_hint(dst, my, 0, yrow, z, BAR(LB_FULL + slot), pol_stream);
+                for (int c = 0; c < nch; ++c)
+                    tma_load_3d_hint(dst + (uint32_t)((1 + c) * HSLOT), mp, 0, prow + c * 128, z, BAR(LB_FULL + slot), pol_keep);
             }
             __syncwarp();
             ++g;
@@ -344,12 +422,13 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
         };
         for (int64_t i = 0; i < ntl && ok; ++i) {
             const int32_t row0 = (int32_t)((blockIdx.x + i * gridDim.x) * WIDE_TILE);
-            for (int gq = 0; gq < NG && ok; ++gq) {
+            for (int t = 0; t < nsteps && ok; ++t) {
+                const int gq = step_group(t);
                 const int nch = (NC - 2 * gq < 2) ? (NC - 2 * gq) : 2;
+                const bool hi_only = leading_only(gq);
                 for (int z = 0; z < NZ && ok; ++z) {
-                    const bool hi_only = gq >= p.hi_group && gq < p.hi_end;
-                    ok = item(&tm_yhi, &tm_ylo, row0, z, false, hi_only);
-                    for (int c = 0; c < nch && ok; ++c) ok = item(&tm_phi, &tm_plo, (2 * gq + c) * 128, z, true, hi_only);
+                    ok = stage(&tm_yhi, &tm_phi, row0, 2 * gq * 128, nch, z);
+                    if (ok && !hi_only) ok = stage(&tm_ylo, &tm_plo, row0, 2 * gq * 128, nch, z);
                 }
             }
         }
@@ -362,7 +441,7 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
         }
     } else {
         // =========================== MMA warp ===========================
-        const uint32_t idesc = make_idesc(WIDE_TILE, 128, 0);
+        const uint32_t idesc1 = make_idesc(WIDE_TILE, 128, 0), idesc2 = make_idesc(WIDE_TILE, 256, 0);
         const uint64_t d0 = make_desc(smem_u32(smem), 16, 1024);
         bool alive = true;
         auto wait_all = [&](uint32_t bar, uint32_t parity) -> bool {
@@ -373,41 +452,60 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
             return ok != 0u;
         };
         int64_t g = 0;
-        uint32_t groups_done = 0;
+        uint32_t ub0 = 0, ub1 = 0;                           // uses of the two accumulator halves
+        int nb = 0;
+        auto take = [&](int& slot) -> bool {                 // the next stage of the ring, once it has landed
+            slot = (int)(g % L_SLOTS);
+            const bool ok = wait_all(BAR(LB_FULL + slot), (uint32_t)((g / L_SLOTS) & 1));
+            ++g;
+            return ok;
+        };
         for (int64_t i = 0; i < ntl && alive; ++i) {
-            for (int gq = 0; gq < NG && alive; ++gq) {
+            for (int t = 0; t < nsteps && alive; ++t) {
+                const int gq = step_group(t);
                 const int nch = (NC - 2 * gq < 2) ? (NC - 2 * gq) : 2;
-                if (groups_done > 0 && !wait_all(BAR(LB_LEMPTY), (groups_done - 1) & 1u)) { alive = false; break; }
-                for (int z = 0; z < NZ && alive; ++z) {
-                    const int sy = (int)(g % L_SLOTS);
-                    if (!wait_all(BAR(LB_FULL + sy), (uint32_t)((g / L_SLOTS) & 1))) { alive = false; break; }
-                    ++g;
-                    for (int c = 0; c < nch; ++c) {
-                        const int sp = (int)(g % L_SLOTS);
-                        if (!wait_all(BAR(LB_FULL + sp), (uint32_t)((g / L_SLOTS) & 1))) { alive = false; break; }
-                        ++g;
-                        if (elect_one()) {
-                            const uint64_t ah = d0 + ((sy * SLOT) >> 4), al = ah + ((SLOT / 2) >> 4);
-                            const uint64_t bh = d0 + ((sp * SLOT) >> 4), bl = bh + ((SLOT / 2) >> 4);
-                            const uint32_t d = tmem + c * 128, dc = tmem + 256 + c * 128;
-                            // the two small cross products into their own accumulator, the leading product into the main one:
-                            // the same three chains, in the same order, as the E-step of sweep 2
-                            if (!(gq >= p.hi_group && gq < p.hi_end)) {
-#pragma unroll
-                                for (int j = 0; j < 4; ++j) mma_ss(dc, ah + ((j * 32) >> 4), bl + ((j * 32) >> 4), idesc, (z > 0 || j > 0) ? 1u : 0u);
-#pragma unroll
-                                for (int j = 0; j < 4; ++j) mma_ss(dc, al + ((j * 32) >> 4), bh + ((j * 32) >> 4), idesc, 1u);
-                            }
-#pragma unroll
-                            for (int j = 0; j < 4; ++j) mma_ss(d, ah + ((j * 32) >> 4), bh + ((j * 32) >> 4), idesc, (z > 0 || j > 0) ? 1u : 0u);
-                            mma_commit(BAR(LB_EMPTY + sp));
-                            if (c == nch - 1) mma_commit(BAR(LB_EMPTY + sy));
-                            if (c == nch - 1 && z == NZ - 1) mma_commit(BAR(LB_LFULL));
-                        }
-                        __syncwarp();
-                    }
+                const bool hi_only = leading_only(gq);
+                const uint32_t idesc = nch == 2 ? idesc2 : idesc1;       // both chunks of the group as one operand of 256 rows
+                // the softmax warps must be done with the accumulator columns this group writes
+                int half = 0;
+                if (hi_only) {
+                    half = nb;
+                    nb ^= 1;
+                    const uint32_t u = half ? ub1 : ub0;
+                    if (u > 0 && !wait_all(BAR(LB_LEMPTY + half), (u - 1) & 1u)) { alive = false; break; }
+                } else {
+                    if (ub0 > 0 && !wait_all(BAR(LB_LEMPTY), (ub0 - 1) & 1u)) { alive = false; break; }
+                    if (ub1 > 0 && !wait_all(BAR(LB_LEMPTY + 1), (ub1 - 1) & 1u)) { alive = false; break; }
                 }
-                ++groups_done;
+                const uint32_t d = tmem + half * 256, dc = tmem + 256;
+                for (int z = 0; z < NZ && alive; ++z) {
+                    int sh = 0, sl = 0;
+                    if (!take(sh)) { alive = false; break; }
+                    if (!hi_only && !take(sl)) { alive = false; break; }
+                    if (elect_one()) {
+                        const uint64_t ah = d0 + ((sh * L_STAGE) >> 4), bh = ah + (HSLOT >> 4);
+                        // the two small cross products into their own accumulator, the leading product into the main one:
+                        // the same three chains, in the same order, as the E-step of sweep 2
+                        if (!hi_only) {
+                            const uint64_t al = d0 + ((sl * L_STAGE) >> 4), bl = al + (HSLOT >> 4);
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) mma_ss(dc, ah + ((j * 32) >> 4), bl + ((j * 32) >> 4), idesc, (z > 0 || j > 0) ? 1u : 0u);
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) mma_ss(dc, al + ((j * 32) >> 4), bh + ((j * 32) >> 4), idesc, 1u);
+                        }
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) mma_ss(d, ah + ((j * 32) >> 4), bh + ((j * 32) >> 4), idesc, (z > 0 || j > 0) ? 1u : 0u);
+                        mma_commit(BAR(LB_EMPTY + sh));
+                        if (!hi_only) mma_commit(BAR(LB_EMPTY + sl));
+                        if (z == NZ - 1) {
+                            if (hi_only) mma_commit(BAR(LB_LFULL + half));
+                            else { mma_commit(BAR(LB_LFULL)); mma_commit(BAR(LB_LFULL + 1)); }
+                        }
+                    }
+                    __syncwarp();
+                }
+                if (hi_only) { if (half) ++ub1; else ++ub0; }
+                else { ++ub0; ++ub1; }
             }
         }
         if (elect_one()) mma_commit(BAR(LB_FINAL));
@@ -2128,7 +2226,7 @@ cudaError_t launch_transform_wide(cudaStream_t s, const float* X, int64_t n, int
 }
 
 cudaError_t launch_lse_wide(cudaStream_t s, int64_t n, int D, int K, int Kg, int n_listed, int n_slots, const WideBuffers& wb,
-                            int num_sms, int* status, int ntop, int hi_first_slots) {
+                            int num_sms, int* status, int ntop, int hi_first_slots, bool pre_pass) {
     if (n < 1 || n > WIDE_PIECE || Kg < 0 || Kg > K || (Kg < 1 && n_listed < 1)) return cudaErrorInvalidValue;
     const WidePlan pl = wide_plan(D, K, num_sms);
     const int64_t rp = rows_padded_of(n);
@@ -2156,8 +2254,11 @@ cudaError_t launch_lse_wide(cudaStream_t s, int64_t n, int D, int K, int Kg, int
     p.scr = reinterpret_cast<const float2*>(wb.scr);
     p.scr_e = wb.scr_e; p.scr_mask = wb.scr_mask; p.slot_of = wb.slot_of; p.n2 = wb.n2; p.cand = wb.cand;
     p.cand_words = (n_slots + 31) / 32; p.scr_group = Kgp / 256; p.ctl = wb.ctl;
-    p.hi_group = 0x7fffffff; p.hi_end = 0x7fffffff;
-    if (ntop == 2 && screen && hi_first_slots >= 0) p.hi_group = (Kgp + hi_first_slots + 255) / 256;        // the EM step's screening mode
+    p.hi_group = 0x7fffffff; p.hi_end = 0x7fffffff; p.pre_pass = 0;
+    if (ntop == 2 && screen && hi_first_slots >= 0) {                                                      // the EM step's screening mode
+        p.hi_group = (Kgp + hi_first_slots + 255) / 256;
+        p.pre_pass = pre_pass ? 1 : 0;
+    }
     if (ntop != 2 && hi_first_slots >= 0) { p.hi_group = 0; p.hi_end = Kgp / 256; }                         // the assignment's evaluated groups
     const int64_t ntiles = (n + WIDE_TILE - 1) / WIDE_TILE;
     const unsigned grid = (unsigned)(ntiles < num_sms ? ntiles : num_sms);

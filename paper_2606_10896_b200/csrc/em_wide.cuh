@@ -116,7 +116,9 @@ cudaError_t launch_cand_count_wide(cudaStream_t s, const WideBuffers& wb);
 // hi_first_slots >= 0 (with parameters prepared in hi_mode): the slots of the list's first kind (flags[5]); the groups of
 // 256 positions behind them are screened by the leading product alone.
 cudaError_t launch_lse_wide(cudaStream_t s, int64_t n, int D, int K, int Kg, int n_listed, int n_slots, const WideBuffers& wb,
-                            int num_sms, int* status, int ntop = 2, int hi_first_slots = -1);
+                            int num_sms, int* status, int ntop = 2, int hi_first_slots = -1, bool pre_pass = false);
+// pre_pass (with hi_first_slots >= 0): every tile first sweeps those groups once for the largest lower bound alone, so that
+// the screening threshold is final before anything is marked.
 // Top-m assignment of the n points of a piece from what launch_lse_wide (ntop >= m + 2; screened: it also marked the listed
 // pairs) and launch_norm_wide left in wb: idx [n][m], resp [n][m] (may be NULL); rows whose answer is not certain are appended to unc_rows
 // (unc_count += 1 each) and left unwritten.  mu, w2, c2d: the FP32 path's derived parameters.

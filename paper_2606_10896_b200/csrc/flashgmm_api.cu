@@ -181,8 +181,9 @@ struct gmm_ctx {
     int wide_mode = 0;               // GMM_WIDE_MODE: 0 = automatic, 1 = "sweeps" (two tensor sweeps, few components exact),
                                      // 2 = "screen" (one tensor sweep screens every pair, every component evaluated exactly)
     double wide_probe_limit = 0.0;   // automatic mode: "screen" while a sample of the points has at most this many marked pairs per
-                                     // point (0: K D / 70000, or K D / 8192 below 128 points per component)
+                                     // point (0: K / 400, or K / 24 below 128 points per component)
     bool wide_screen_all = false;    // the current step runs in "screen" mode
+    bool wide_pre = true;            // GMM_WIDE_PRE=0: no first pass for the screening threshold
     bool wide_hi = true;             // GMM_WIDE_HI=0: the screening mode forms all three products for every component
     int wide_sparse = 1;             // GMM_WIDE_SPARSE: 0 = the listed components always go through the dense FP32 kernels,
                                      // 1 = pair by pair unless sweep 1 marks too many pairs, 2 = always pair by pair (tests)
@@ -446,13 +447,14 @@ int prepare_and_choose(gmm_ctx* ctx, int64_t N, int D, int K, const float* pi, c
         int fl[8];
         const bool can_probe = Xprobe != nullptr && n_probe >= 1;
         // Automatic choice, step by step: the screening sweep is tried on the first 8192 rows, and "screen" is taken if it marks
-        // few enough pairs per point.  A marked pair costs about 1.3 ns (exact evaluation) and a kept one 5 ns more (its
-        // statistics); what "screen" saves is the second tensor sweep, K D / 50 ps per point (60 ns at config 5's shape), so
-        // from 128 points per component on the limit is K D / 70000 marked pairs per point - config 5: 45, which its first
-        // three iterations from a data-row initialisation exceed (74, 97, 71 at N = 1M: 180-300 ms per million points
-        // against 122 for "sweeps") and the later ones do not (26 at N = 1M: 82 ms against 101; 37-42 at N = 10M: 89-96
-        // against 105).  Below 128 points per component "sweeps" is no
-        // alternative (it would list most components as light) and the FP32 kernels cost K D / 2 ns per point: K D / 8192.
+        // few enough pairs per point.  With the threshold final before anything is marked, nearly every marked pair is kept,
+        // and a kept pair costs 4-7 ns at D = 768 (exact evaluation plus its statistics: measured 43-76 ms per 10 million
+        // points and pair per point).  What "screen" saves is the second tensor sweep, whose cost per point grows with K D
+        // like the pair's does with D: from 128 points per component on the limit is K / 400 marked pairs per point
+        // (config 5: 10; its iterations from a data-row initialisation mark 9, 30, 11, 4.6, 3.3 and take 0.88, 2.05, 0.96,
+        // 0.72, 0.68 s in "screen" against 1.24, 1.28, 1.04, 1.06, 1.06 s in "sweeps").  Below 128 points per component
+        // "sweeps" is no alternative (it would list most components as light) and the FP32 kernels cost K D / 2 ns per
+        // point: K / 24.
         const bool few_points = N < WIDE_AUTO_MIN_POINTS_PER_COMPONENT * K;
         if (ctx->wide_mode == 2 || (ctx->wide_mode == 0 && can_probe)) {
             KL(launch_prepare_wide(ctx->stream, D, K, pi, mu, var, wb, limit, INFINITY, ctx->wide_hi ? 1 : 0));      // every component is listed
@@ -468,11 +470,11 @@ int prepare_and_choose(gmm_ctx* ctx, int64_t N, int D, int K, const float* pi, c
                 CU(launch_cand_clear_wide(ctx->stream, np, n_list, wb));
                 KL(launch_norm_wide(ctx->stream, Xprobe, np, D, wb));
                 KL(launch_transform_wide(ctx->stream, Xprobe, np, D, wb, &ctx->result()->status));
-                KL(launch_lse_wide(ctx->stream, np, D, K, fl[6], fl[4], n_list, wb, ctx->sms, &ctx->result()->status, 2, ctx->wide_hi ? fl[5] : -1));
+                KL(launch_lse_wide(ctx->stream, np, D, K, fl[6], fl[4], n_list, wb, ctx->sms, &ctx->result()->status, 2, ctx->wide_hi ? fl[5] : -1, ctx->wide_pre));
                 int marks = 0;
                 CU(cudaMemcpyAsync(&marks, wb.ctl, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
                 CU(cudaStreamSynchronize(ctx->stream));
-                const double auto_limit = (double)n_list * D / (few_points ? 8192.0 : 70000.0);
+                const double auto_limit = (double)n_list / (few_points ? 24.0 : 400.0);
                 ok = (double)marks <= (ctx->wide_probe_limit > 0.0 ? ctx->wide_probe_limit : auto_limit) * (double)np;
             }
             if (ok) {
@@ -574,7 +576,7 @@ int accumulate_points(gmm_ctx* ctx, int path, const float* X, int64_t n, int D, 
             CHECK(prof_begin(ctx));
             KL(launch_transform_wide(ctx->stream, Xs, cnt, D, wb, &ctx->result()->status));
             KL(launch_lse_wide(ctx->stream, cnt, D, K, Kg, screen ? n_listed : 0, n_ill, wb, ctx->sms, &ctx->result()->status, 2,
-                               (all && ctx->wide_hi) ? ctx->wide_n_first : -1));
+                               (all && ctx->wide_hi) ? ctx->wide_n_first : -1, ctx->wide_pre));
             if (ctx->wide_refine && !all) KL(launch_refine_wide(ctx->stream, Xs, cnt, D, K, mu, ctx->w2(), ctx->c2d(), wb));
             else CU(cudaMemcpyAsync(wb.logz_x, wb.logz, (size_t)cnt * 8, cudaMemcpyDeviceToDevice, ctx->stream));
             if (n_ill > 0) {
@@ -582,7 +584,7 @@ int accumulate_points(gmm_ctx* ctx, int path, const float* X, int64_t n, int D, 
                     // more than one pair in 64 marked (or the pair-by-pair route switched off): the dense kernels are cheaper
                     // ("screen" mode: the dense alternative evaluates every component, so the pair route pays for longer)
                     const long long max_pairs = ctx->wide_sparse >= 2 ? ((long long)1 << 62)
-                                              : all ? (long long)((double)cnt * n_ill * D / 8192.0) : (long long)cnt * n_ill / 64;
+                                              : all ? (long long)cnt * n_ill / 24 : (long long)cnt * n_ill / 64;
                     KL(launch_cand_gate_wide(ctx->stream, wb, max_pairs));
                     KL(launch_cand_lse_wide(ctx->stream, Xs, cnt, D, n_ill, wb, ctx->logZ2()));
                 }
@@ -728,6 +730,7 @@ int gmm_create(gmm_ctx** out, int device, void* cuda_stream) {
     if (const char* e = std::getenv("GMM_WIDE_REFINE")) ctx->wide_refine = std::atoi(e) != 0;
     if (const char* e = std::getenv("GMM_WIDE_SPARSE")) ctx->wide_sparse = std::atoi(e);
     if (const char* e = std::getenv("GMM_WIDE_HI")) ctx->wide_hi = std::atoi(e) != 0;
+    if (const char* e = std::getenv("GMM_WIDE_PRE")) ctx->wide_pre = std::atoi(e) != 0;
     if (const char* e = std::getenv("GMM_WIDE_MODE")) ctx->wide_mode = !std::strcmp(e, "sweeps") ? 1 : !std::strcmp(e, "screen") ? 2 : 0;
     if (const char* e = std::getenv("GMM_WIDE_PROBE_LIMIT")) ctx->wide_probe_limit = std::atof(e);
     if (const char* e = std::getenv("GMM_WIDE_PIECE")) {

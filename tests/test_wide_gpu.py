@@ -129,8 +129,8 @@ def test_wide_auto_path_rule(fg, ctx):
     ctx.gmm_set_path(fg.GMM_PATH_AUTO)
     ctx.gmm_em_step(_t(X), _t(pi), _t(mu), _t(var))
     assert ctx.gmm_last_path() == fg.GMM_PATH_TENSOR and ctx.gmm_last_exact_count() == 0
-    ctx.gmm_em_step(_t(X[:100 * K]), _t(pi), _t(mu), _t(var))
-    assert ctx.gmm_last_path() == fg.GMM_PATH_FP32       # (K = 64, D = 256: only 2 marked pairs per point would pay)
+    _step_and_check(fg, ctx, X[:100 * K], pi, mu, var, "100 points per component, separate clusters")
+    assert ctx.gmm_last_path() == fg.GMM_PATH_TENSOR and ctx.gmm_last_exact_count() == K      # (one marked pair per point)
     K2, D2 = 1024, 512
     X2, pi2, mu2, var2 = _clustered(np.random.default_rng(15), 40 * K2, D2, K2)
     with fg.Context(0) as c2:

@@ -399,7 +399,11 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
         // the leading product only) the lo planes' stage.
         int64_t g = 0;
         bool ok = true;
-        const uint64_t pol_keep = l2_policy_evict_last(), pol_stream = l2_policy_evict_first();
+        // Both streams are kept in L2 with priority: the coefficient atoms are read by every CTA for every tile, the tile's
+        // own atoms once per step of the tile.  (Marked evict-first, the tile's atoms missed L2 on nearly every re-read -
+        // a third of the sweep's sectors came from DRAM, 17 % of its time: L2 is full of older lines of normal priority,
+        // e.g. the planes as the transform wrote them, which such lines do not displace.)
+        const uint64_t pol_keep = l2_policy_evict_last();
         auto stage = [&](const CUtensorMap* my, const CUtensorMap* mp, int32_t yrow, int32_t prow, int nch, int32_t z) -> bool {
             const int slot = (int)(g % L_SLOTS);
             const int64_t use = g / L_SLOTS;
@@ -411,8 +415,7 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
             if (elect_one()) {
                 const uint32_t dst = smem_u32(smem + slot * L_STAGE);
                 bar_expect_tx(BAR(LB_FULL + slot), (uint32_t)((1 + nch) * HSLOT));
-                // the coefficient atoms are read by every CTA for every tile, the tile's own atoms once per group
-                tma_load_3d_hint(dst, my, 0, yrow, z, BAR(LB_FULL + slot), pol_stream);
+                tma_load_3d_hint(dst, my, 0, yrow, z, BAR(LB_FULL + slot), pol_keep);
                 for (int c = 0; c < nch; ++c)
                     tma_load_3d_hint(dst + (uint32_t)((1 + c) * HSLOT), mp, 0, prow + c * 128, z, BAR(LB_FULL + slot), pol_keep);
             }

@@ -181,7 +181,7 @@ struct gmm_ctx {
     int wide_mode = 0;               // GMM_WIDE_MODE: 0 = automatic, 1 = "sweeps" (two tensor sweeps, few components exact),
                                      // 2 = "screen" (one tensor sweep screens every pair, every component evaluated exactly)
     double wide_probe_limit = 0.0;   // automatic mode: "screen" while a sample of the points has at most this many marked pairs per
-                                     // point (0: K / 400, or K / 24 below 128 points per component)
+                                     // point (0: K / 300, or K / 24 below 128 points per component)
     bool wide_screen_all = false;    // the current step runs in "screen" mode
     bool wide_pre = true;            // GMM_WIDE_PRE=0: no first pass for the screening threshold
     bool wide_hi = true;             // GMM_WIDE_HI=0: the screening mode forms all three products for every component
@@ -474,7 +474,7 @@ int prepare_and_choose(gmm_ctx* ctx, int64_t N, int D, int K, const float* pi, c
                 int marks = 0;
                 CU(cudaMemcpyAsync(&marks, wb.ctl, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
                 CU(cudaStreamSynchronize(ctx->stream));
-                const double auto_limit = (double)n_list / (few_points ? 24.0 : 400.0);
+                const double auto_limit = (double)n_list / (few_points ? 24.0 : 300.0);
                 ok = (double)marks <= (ctx->wide_probe_limit > 0.0 ? ctx->wide_probe_limit : auto_limit) * (double)np;
             }
             if (ok) {

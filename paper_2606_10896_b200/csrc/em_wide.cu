@@ -1465,7 +1465,8 @@ __global__ void __launch_bounds__(256, 4) wide_cand_lse_kernel(const float* __re
                                                             const float* __restrict__ mu_c, const float* __restrict__ w2_c,
                                                             const double* __restrict__ c2d_c, const double* __restrict__ logz,
                                                             double* __restrict__ out, int* __restrict__ ctl,
-                                                            int* __restrict__ slot_cnt) {
+                                                            int* __restrict__ slot_cnt, float* __restrict__ pair_val,
+                                                            int* __restrict__ pair_off, double* __restrict__ pair_best) {
     if (ctl[1] != 0) return;
     __shared__ double lbuf[8][CAND_KEEP];
     __shared__ unsigned short slist[8][CAND_LIST];
@@ -1617,6 +1618,15 @@ __global__ void __launch_bounds__(256, 4) wide_cand_lse_kernel(const float* __re
     }
     __syncwarp();
     const bool listed = total <= CAND_LIST;                   // (else: the row is scanned word by word, as a fallback)
+    // Room for the exact values of the point's pairs (the statistics kernel reads them back instead of evaluating its pairs
+    // again).  Where the room starts depends on timing, what is stored there does not.  No room left: ctl[5] tells the
+    // statistics kernel to evaluate every pair of the piece itself.
+    int off = -1;
+    if (lane == 0) {
+        off = atomicAdd(ctl + 4, total);
+        if (off < 0 || off > WIDE_PAIR_VALS - total) { off = -1; ctl[5] = 1; }
+    }
+    off = __shfl_sync(0xffffffffu, off, 0);
     double best = logz[i];
     int idx = 0;
     {
@@ -1671,6 +1681,7 @@ __global__ void __launch_bounds__(256, 4) wide_cand_lse_kernel(const float* __re
             if (lane == 0) {
                 atomicOr(candT + (size_t)slot * WIDE_CANDT_WORDS + (i >> 5), 1u << (i & 31));
                 atomicAdd(slot_cnt + slot, 1);
+                if (off >= 0) pair_val[off + at] = (float)(l - best);       // in [-40, 0]
             }
             ++kept;
         }
@@ -1692,15 +1703,19 @@ __global__ void __launch_bounds__(256, 4) wide_cand_lse_kernel(const float* __re
     if (lane == 0) {
         out[i] = kept ? m + log2(ssum) : -CUDART_INF;
         if (kept) atomicAdd(ctl + 3, kept);
+        pair_off[i] = off;
+        pair_best[i] = best;
     }
 }
 
 // One block per slot: the points marked for it in the transposed map, in ascending order (the order of the additions is
 // fixed: same bits in every run).  The block lists its points in shared memory (up to MS_CAP per pass over the map), then
-// takes them eight at a time: every thread loads its 3-4 dimensions of the eight rows (all loads in flight together), the
-// eight quadratic forms are reduced over the block (fp32 per thread, float64 from there), r = 2^(log2 z - log2 Z), and every
-// thread adds r (x - g), r (x - g)^2 for its dimensions in float64.  The sums are shifted back to the origin and added to
-// the slot's statistics.
+// looks up each pair's exact log2 z as wide_cand_lse_kernel left it (the pair's rank among the point's marked pairs = bits
+// below the slot in the point's row of the map) and takes the points eight at a time: every thread loads its 3-4
+// dimensions of the eight rows (all loads in flight together) and adds r (x - g), r (x - g)^2, r = 2^(log2 z - log2 Z),
+// for its dimensions in float64.  Without the stored values (a piece with more marked pairs than there is room for) the
+// eight quadratic forms are evaluated again and reduced over the block (fp32 per thread, float64 from there).  The sums
+// are shifted back to the origin and added to the slot's statistics.
 constexpr int MS_CAP = 1024, MS_B = 8;
 constexpr int MS_SEG = WIDE_HEAVY_SEG;     // a component kept for many points of a piece is split over this many blocks ...
 constexpr int MS_SPLIT_MIN = 512;         // ... from this many pairs on
@@ -1741,8 +1756,12 @@ __global__ void __launch_bounds__(256) wide_cand_mstep_kernel(const float* __res
                                                               const float* __restrict__ gd, const double* __restrict__ logz_x,
                                                               double* __restrict__ Nk_c, double* __restrict__ S1_c,
                                                               double* __restrict__ S2_c, const int* __restrict__ ctl,
-                                                              const int* __restrict__ heavy_of, double* __restrict__ heavy_part) {
+                                                              const int* __restrict__ heavy_of, double* __restrict__ heavy_part,
+                                                              const unsigned* __restrict__ cand, int cand_words,
+                                                              const float* __restrict__ pair_val, const int* __restrict__ pair_off,
+                                                              const double* __restrict__ pair_best) {
     if (ctl[1] != 0) return;
+    const bool stored = ctl[5] == 0;                         // the pairs' exact values are there
     const int slot = blockIdx.x, seg = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (list[slot] < 0) return;
     const int hv = heavy_of[slot];
@@ -1762,6 +1781,7 @@ __global__ void __launch_bounds__(256) wide_cand_mstep_kernel(const float* __res
         cnt += __popc(mine[j]);
     }
     __shared__ int rows_s[MS_CAP];
+    __shared__ double r_s[MS_CAP];
     __shared__ int wtot[8];
     __shared__ double red_s[8][MS_B];
     int incl = cnt;
@@ -1806,6 +1826,46 @@ __global__ void __launch_bounds__(256) wide_cand_mstep_kernel(const float* __res
         }
         __syncthreads();
         const int here = (total - base < MS_CAP) ? (total - base) : MS_CAP;
+        if (stored) {
+            for (int e = tid; e < here; e += 256) {
+                const int row = rows_s[e];
+                const unsigned* cr = cand + (size_t)row * cand_words;
+                int rank = 0;
+                for (int w = 0; w < (slot >> 5); ++w) rank += __popc(__ldg(cr + w));
+                rank += __popc(__ldg(cr + (slot >> 5)) & ((1u << (slot & 31)) - 1u));
+                const int off = pair_off[row];
+                r_s[e] = exp2((double)pair_val[off + rank] + (pair_best[row] - logz_x[row]));
+            }
+            __syncthreads();
+            for (int e0 = 0; e0 < here; e0 += MS_B) {
+                float xv[MS_B][4];
+#pragma unroll
+                for (int b = 0; b < MS_B; ++b) {
+                    const bool in = e0 + b < here;
+                    const float* xr = X + (size_t)(in ? rows_s[e0 + b] : rows_s[e0]) * D;
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const int d = tid + 256 * q;
+                        xv[b][q] = (d < D) ? __ldg(xr + d) : 0.f;
+                    }
+                }
+#pragma unroll
+                for (int b = 0; b < MS_B; ++b) {
+                    if (e0 + b < here) {                     // block-uniform
+                        const double r = r_s[e0 + b];
+                        nk += r;
+#pragma unroll
+                        for (int qq = 0; qq < 4; ++qq) {
+                            const double xd = (double)(xv[b][qq] - g_r[qq]);
+                            s1[qq] += r * xd;
+                            s2[qq] += r * xd * xd;
+                        }
+                    }
+                }
+            }
+            __syncthreads();                                 // rows_s, r_s are rewritten by the next pass
+            continue;
+        }
         for (int e0 = 0; e0 < here; e0 += MS_B) {
             float xv[MS_B][4];
             float part[MS_B];
@@ -2181,7 +2241,7 @@ cudaError_t launch_cand_lse_wide(cudaStream_t s, const float* X, int64_t n, int 
                                  double* logz_ill) {
     const int words = (n_slots + 31) / 32;
     wide_cand_lse_kernel<<<(unsigned)((n + 7) / 8), 256, 0, s>>>(X, n, D, words, wb.cand, wb.candT, wb.mu_c, wb.w2_c, wb.c2d_c, wb.logz,
-                                                                 logz_ill, wb.ctl, wb.slot_cnt);
+                                                                 logz_ill, wb.ctl, wb.slot_cnt, wb.pair_val, wb.pair_off, wb.pair_best);
     return cudaGetLastError();
 }
 
@@ -2193,7 +2253,8 @@ cudaError_t launch_cand_mstep_wide(cudaStream_t s, const float* X, int64_t n, in
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     wide_cand_mstep_kernel<<<dim3((unsigned)n_slots, MS_SEG), 256, 0, s>>>(X, n, D, wb.ill_list, wb.candT, wb.mu_c, wb.w2_c, wb.c2d_c, wb.gd,
-                                                                        wb.logz_x, Nk_c, S1_c, S2_c, wb.ctl, wb.heavy_of, wb.heavy_part);
+                                                                        wb.logz_x, Nk_c, S1_c, S2_c, wb.ctl, wb.heavy_of, wb.heavy_part,
+                                                                        wb.cand, (n_slots + 31) / 32, wb.pair_val, wb.pair_off, wb.pair_best);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     wide_heavy_combine_kernel<<<MS_HEAVY, 256, 0, s>>>(D, wb.heavy_slot, wb.heavy_part, Nk_c, S1_c, S2_c, wb.ctl);

@@ -12,6 +12,8 @@ constexpr int WIDE_MAX_K = 4096;
 constexpr int64_t WIDE_PIECE = 1 << 17;      // points per pair of launches: capacity of the fp16 planes of Y in scratch
 constexpr int WIDE_BATCH = 256;              // points per batch of the second sweep
 constexpr int WIDE_TILE = 128;               // points per tile of the first sweep
+constexpr int WIDE_PAIR_VALS = 32 * (int)WIDE_PIECE; // exact values kept from the pairs' evaluation for their statistics (more marked
+                                                // pairs in a piece: the statistics kernel evaluates its pairs again)
 constexpr int WIDE_MAX_ILL = WIDE_MAX_K + 64; // slots of the list of components evaluated exactly (all of them may be; + the gap)
 constexpr int WIDE_LL_BLOCKS = 64;           // per-block partial sums of the log-likelihood
 constexpr int WIDE_MAX_TOP = 10;             // candidates per point sweep 1 can report (the top-m assignment asks for m + 2)
@@ -75,6 +77,10 @@ struct WideBuffers {
     int* heavy_of;  // [slots] index of a slot's partial sums when its points are split over several blocks, else -1
     int* heavy_slot;// [WIDE_HEAVY_SLOTS] the slot of each set of partial sums, -1 if unused
     double* heavy_part;    // [WIDE_HEAVY_SLOTS][WIDE_HEAVY_SEG][1 + 2 D] partial (N_k, S1, S2) of the split slots' segments
+    float* pair_val;   // [WIDE_PAIR_VALS] exact log2 z of a piece's kept pairs relative to the point's best value, a point's
+                       // marked pairs consecutive and in slot order (positions from a counter: ctl[4])
+    int* pair_off;     // [WIDE_PIECE] where a point's values start
+    double* pair_best; // [WIDE_PIECE] the point's best value (the reference of its pair_val entries)
     int* ctl;       // [8]: [0] pairs sweep 1 let through, [1] nonzero: too many, the FP32 kernels evaluate the sub-mixture
                     //      densely, [2] nonzero: the pairs are evaluated one by one, [3] pairs that mattered
 };

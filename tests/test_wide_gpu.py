@@ -173,6 +173,20 @@ def test_wide_screen_mode_against_oracle(fg, monkeypatch, N, D, K):
             assert np.array_equal(u, v.cpu().numpy())
 
 
+def test_wide_screen_mode_more_pairs_than_stored_values(fg, monkeypatch):
+    """Clusters on top of each other, every pair marked: more marked pairs in a piece (40,000 x 130) than the buffer of exact
+    pair values holds (32 x 2^17), so the statistics kernel evaluates its pairs itself."""
+    monkeypatch.setenv("GMM_WIDE_MODE", "screen")
+    monkeypatch.setenv("GMM_WIDE_SPARSE", "2")
+    N, D, K = 40_000, 200, 130
+    X, pi, mu, var = _clustered(np.random.default_rng(77), N, D, K, sep=0.01)
+    with fg.Context(0) as c:
+        c.gmm_set_path(fg.GMM_PATH_TENSOR)
+        _step_and_check(fg, c, X, pi, mu, var, "every pair marked")
+        marked, kept, dense = c.gmm_last_exact_pairs()
+        assert dense == 0 and marked > 32 * 2 ** 17 and kept > N
+
+
 def test_wide_screen_mode_free_running_fit(fg, monkeypatch):
     monkeypatch.setenv("GMM_WIDE_MODE", "screen")
     rng = np.random.default_rng(19)

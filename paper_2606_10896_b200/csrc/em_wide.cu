@@ -93,6 +93,9 @@ struct LseParams {
     int scr_group;       // first group of 256 columns that holds listed components (they hold nothing else from there on)
     int hi_group;        // groups [hi_group, hi_end): only the leading product (Y_hi P_hi) is formed, with wider allowances
     int hi_end;
+    unsigned* rec;       // NULL, or [n][WIDE_REC]: the marks' upper bounds, for the filter that follows
+    int* rec_cnt;        // [n]
+    float* rec_thr;      // [n] the point's final threshold
     int pre_pass;        // 1: before a tile's sweep proper, the groups from hi_group on are swept once for their lower bounds only
     int* ctl;
 };
@@ -138,6 +141,7 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
     // slower warps may still read the other): (t, c, screening offset, screening slope), the allowance alone, the chunk masks.
     // Read from global memory inside the loops over the accumulators they cost a trip to L2 per pair of components (the
     // shared-memory ring leaves almost no L1).
+    __shared__ int rcnt_s[128];                          // marks of the tile's points so far
     __shared__ float4 tab_s[2][2][128];
     __shared__ float tabe_s[2][2][128];
     __shared__ int tabm_s[2][2][4];
@@ -156,6 +160,7 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
 
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L_BAR);
     auto BAR = [&](int i) { return smem_u32(&bars[i]); };
+    if (tid < 128) rcnt_s[tid] = 0;
     if (tid == 0) {
         abort_s = 0;
         drain_s = 0;
@@ -211,6 +216,18 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
             int nhit = 0;
             WideTop<NTOP> tl;                                // the largest logits of this thread's chunks, and where
             tl.init();
+            // A pair that can matter: its bit in the map, and (for the filter that follows the sweep) its upper bound, rounded
+            // up to the 19 bits that share a word with the slot.
+            auto mark = [&](float u, int col) {
+                const int sl = __ldg(p.slot_of + col);
+                if (sl < 0) return;
+                atomicOr(p.cand + row * p.cand_words + (sl >> 5), 1u << (sl & 31));
+                ++nhit;
+                if (p.rec) {
+                    const int ri = atomicAdd(&rcnt_s[pt], 1);
+                    if (ri < WIDE_REC) p.rec[row * WIDE_REC + ri] = (__float_as_uint(u + fabsf(u) * 0.001953125f) & ~0x1FFFu) | (unsigned)sl;
+                }
+            };
             table_load(step_group(0));
             table_store((int)(tcount & 1u));
             for (int t = 0; t < nsteps; ++t) {
@@ -294,14 +311,8 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
                                         thr_base = fmaxf(thr_base, fmaxf(u0 - 2.f * fmaf(sq.y, nrm, se.x), u1 - 2.f * fmaf(sq.w, nrm, se.y)));
                                         const float thr = thr_base - 40.f;
                                         if (ph == 0) continue;                          // (lower bounds only)
-                                        if (!(u0 < thr) && sq.x > -CUDART_INF_F) {
-                                            const int sl = __ldg(p.slot_of + col0 + j);
-                                            if (sl >= 0) { atomicOr(p.cand + row * p.cand_words + (sl >> 5), 1u << (sl & 31)); ++nhit; }
-                                        }
-                                        if (!(u1 < thr) && sq.z > -CUDART_INF_F) {
-                                            const int sl = __ldg(p.slot_of + col0 + j + 1);
-                                            if (sl >= 0) { atomicOr(p.cand + row * p.cand_words + (sl >> 5), 1u << (sl & 31)); ++nhit; }
-                                        }
+                                        if (!(u0 < thr) && sq.x > -CUDART_INF_F) mark(u0, col0 + j);
+                                        if (!(u1 < thr) && sq.z > -CUDART_INF_F) mark(u1, col0 + j + 1);
                                     }
                                 }
                                 continue;
@@ -362,6 +373,7 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
                 if (t + 1 < nsteps) table_store((int)(tcount & 1u));
             }
             // merge the two warpgroups' pairs; warpgroup 0 writes log2 Z and the two leading candidates
+            if (p.rec) xm_s[grp * 128 + pt] = thr_base;      // (each warpgroup's own slot; read after the barrier below)
             if (grp == 1) {
                 merge_s[pt] = make_float2(m_run, s_run);
 #pragma unroll
@@ -381,7 +393,12 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
 #pragma unroll
                     for (int j = 0; j < NTOP; ++j) { tp[j] = tl.a[j]; tp[NTOP + j] = __int_as_float(tl.i[j]); }
                     ll_acc += lz;
+                    if (p.rec) {
+                        p.rec_cnt[row] = rcnt_s[pt];
+                        p.rec_thr[row] = fmaxf(thr_base, xm_s[128 + pt]);
+                    }
                 }
+                rcnt_s[pt] = 0;
             }
             if (nhit > 0) atomicAdd(p.ctl, nhit);
             named_bar_sync(2, 256);                          // merge_s is rewritten by the next tile
@@ -1406,6 +1423,29 @@ __global__ void __launch_bounds__(256) wide_norm_kernel(const float* __restrict_
     if (lane == 0) n2[i] = (s <= 3e38f) ? s : 3e38f;          // (a NaN or an infinity in X is reported by the transform kernel)
 }
 
+// One warp per point: the marks sweep 1 recorded for it, against the point's final threshold.
+__global__ void __launch_bounds__(256) wide_cand_filter_kernel(int64_t n, int words, unsigned* __restrict__ cand,
+                                                               const unsigned* __restrict__ rec, const int* __restrict__ rec_cnt,
+                                                               const float* __restrict__ rec_thr, int* __restrict__ ctl) {
+    const int64_t i = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (i >= n) return;
+    const int cnt = min(rec_cnt[i], WIDE_REC);
+    const float thr = rec_thr[i] - 40.f;
+    int dropped = 0;
+    for (int r = lane; r < cnt; r += 32) {
+        const unsigned v = rec[i * WIDE_REC + r];
+        const int sl = (int)(v & 0x1FFFu);
+        if (__uint_as_float(v & ~0x1FFFu) < thr) {           // (a NaN stays)
+            atomicAnd(cand + i * words + (sl >> 5), ~(1u << (sl & 31)));
+            ++dropped;
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) dropped += __shfl_xor_sync(0xffffffffu, dropped, o);
+    if (lane == 0 && dropped > 0) atomicSub(ctl, dropped);
+}
+
 __global__ void wide_cand_gate_kernel(int* __restrict__ ctl, long long max_pairs) {
     const int dense = ((long long)ctl[0] > max_pairs) ? 1 : 0;
     ctl[1] = dense;
@@ -2227,6 +2267,11 @@ cudaError_t launch_cand_clear_wide(cudaStream_t s, int64_t n, int n_slots, const
     return e;
 }
 
+cudaError_t launch_cand_filter_wide(cudaStream_t s, int64_t n, int n_slots, const WideBuffers& wb) {
+    wide_cand_filter_kernel<<<(unsigned)((n + 7) / 8), 256, 0, s>>>(n, (n_slots + 31) / 32, wb.cand, wb.rec, wb.rec_cnt, wb.rec_thr, wb.ctl);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_cand_gate_wide(cudaStream_t s, const WideBuffers& wb, long long max_pairs) {
     wide_cand_gate_kernel<<<1, 1, 0, s>>>(wb.ctl, max_pairs);
     return cudaGetLastError();
@@ -2290,7 +2335,7 @@ cudaError_t launch_transform_wide(cudaStream_t s, const float* X, int64_t n, int
 }
 
 cudaError_t launch_lse_wide(cudaStream_t s, int64_t n, int D, int K, int Kg, int n_listed, int n_slots, const WideBuffers& wb,
-                            int num_sms, int* status, int ntop, int hi_first_slots, bool pre_pass) {
+                            int num_sms, int* status, int ntop, int hi_first_slots, bool pre_pass, bool record) {
     if (n < 1 || n > WIDE_PIECE || Kg < 0 || Kg > K || (Kg < 1 && n_listed < 1)) return cudaErrorInvalidValue;
     const WidePlan pl = wide_plan(D, K, num_sms);
     const int64_t rp = rows_padded_of(n);
@@ -2319,6 +2364,7 @@ cudaError_t launch_lse_wide(cudaStream_t s, int64_t n, int D, int K, int Kg, int
     p.scr_e = wb.scr_e; p.scr_mask = wb.scr_mask; p.slot_of = wb.slot_of; p.n2 = wb.n2; p.cand = wb.cand;
     p.cand_words = (n_slots + 31) / 32; p.scr_group = Kgp / 256; p.ctl = wb.ctl;
     p.hi_group = 0x7fffffff; p.hi_end = 0x7fffffff; p.pre_pass = 0;
+    p.rec = (record && screen && ntop == 2) ? wb.rec : nullptr; p.rec_cnt = wb.rec_cnt; p.rec_thr = wb.rec_thr;
     if (ntop == 2 && screen && hi_first_slots >= 0) {                                                      // the EM step's screening mode
         p.hi_group = (Kgp + hi_first_slots + 255) / 256;
         p.pre_pass = pre_pass ? 1 : 0;

@@ -14,6 +14,8 @@ constexpr int WIDE_BATCH = 256;              // points per batch of the second s
 constexpr int WIDE_TILE = 128;               // points per tile of the first sweep
 constexpr int WIDE_PAIR_VALS = 32 * (int)WIDE_PIECE; // exact values kept from the pairs' evaluation for their statistics (more marked
                                                 // pairs in a piece: the statistics kernel evaluates its pairs again)
+constexpr int WIDE_REC = 128;                   // marks of a point whose upper bounds sweep 1 records for the filter (more: they stay)
+static_assert(WIDE_MAX_K + 64 <= 8192, "a recorded mark keeps its slot in 13 bits");
 constexpr int WIDE_MAX_ILL = WIDE_MAX_K + 64; // slots of the list of components evaluated exactly (all of them may be; + the gap)
 constexpr int WIDE_LL_BLOCKS = 64;           // per-block partial sums of the log-likelihood
 constexpr int WIDE_MAX_TOP = 10;             // candidates per point sweep 1 can report (the top-m assignment asks for m + 2)
@@ -77,6 +79,9 @@ struct WideBuffers {
     int* heavy_of;  // [slots] index of a slot's partial sums when its points are split over several blocks, else -1
     int* heavy_slot;// [WIDE_HEAVY_SLOTS] the slot of each set of partial sums, -1 if unused
     double* heavy_part;    // [WIDE_HEAVY_SLOTS][WIDE_HEAVY_SEG][1 + 2 D] partial (N_k, S1, S2) of the split slots' segments
+    unsigned* rec;     // [WIDE_PIECE][WIDE_REC] sweep 1's marks of a point: upper bound (rounded up to 19 bits) | slot (13 bits)
+    int* rec_cnt;      // [WIDE_PIECE] how many (may exceed WIDE_REC: the rest was not recorded)
+    float* rec_thr;    // [WIDE_PIECE] the point's final screening threshold (before the 2^-40 margin)
     float* pair_val;   // [WIDE_PAIR_VALS] exact log2 z of a piece's kept pairs relative to the point's best value, a point's
                        // marked pairs consecutive and in slot order (positions from a counter: ctl[4])
     int* pair_off;     // [WIDE_PIECE] where a point's values start
@@ -122,7 +127,10 @@ cudaError_t launch_cand_count_wide(cudaStream_t s, const WideBuffers& wb);
 // hi_first_slots >= 0 (with parameters prepared in hi_mode): the slots of the list's first kind (flags[5]); the groups of
 // 256 positions behind them are screened by the leading product alone.
 cudaError_t launch_lse_wide(cudaStream_t s, int64_t n, int D, int K, int Kg, int n_listed, int n_slots, const WideBuffers& wb,
-                            int num_sms, int* status, int ntop = 2, int hi_first_slots = -1, bool pre_pass = false);
+                            int num_sms, int* status, int ntop = 2, int hi_first_slots = -1, bool pre_pass = false,
+                            bool record = false);
+// record (screening, ntop = 2): every mark's upper bound goes to wb.rec and the point's final threshold to wb.rec_thr, for
+// launch_cand_filter_wide.
 // pre_pass (with hi_first_slots >= 0): every tile first sweeps those groups once for the largest lower bound alone, so that
 // the screening threshold is final before anything is marked.
 // Top-m assignment of the n points of a piece from what launch_lse_wide (ntop >= m + 2; screened: it also marked the listed
@@ -136,6 +144,10 @@ cudaError_t launch_assign_refine_wide(cudaStream_t s, const float* X, int64_t n,
 cudaError_t launch_norm_wide(cudaStream_t s, const float* X, int64_t n, int D, const WideBuffers& wb);
 // Clears wb.ctl, the n rows of wb.cand and the n_slots rows of wb.candT before a piece's first sweep.
 cudaError_t launch_cand_clear_wide(cudaStream_t s, int64_t n, int n_slots, const WideBuffers& wb);
+// After a screening sweep 1 with record = true: the marks whose recorded upper bound lies below the point's final threshold
+// are taken out of wb.cand again and off wb.ctl[0].  (The sweep marks against the threshold as it stands when it meets a
+// pair - the largest lower bound so far - which for most of a point's pairs is far from final.)
+cudaError_t launch_cand_filter_wide(cudaStream_t s, int64_t n, int n_slots, const WideBuffers& wb);
 // After sweep 1: wb.ctl[1] = (wb.ctl[0] > max_pairs), wb.ctl[2] = !wb.ctl[1].
 cudaError_t launch_cand_gate_wide(cudaStream_t s, const WideBuffers& wb, long long max_pairs);
 // The marked pairs evaluated exactly, one warp per point (no-op when wb.ctl[1] is set): logz_ill[i] = log2 of the sum of

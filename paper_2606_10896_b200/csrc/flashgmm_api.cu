@@ -34,7 +34,7 @@ struct ScratchLayout {
     size_t tc_phi, tc_plo, tc_tk, tc_ck, tc_sd, tc_kap, tc_gd, tc_illb, tc_flags, tc_xg, tc_xl, tc_partial, tc_llpart, tc_partial_bytes, tc_yhi, tc_ylo, tc_phirm, tc_plorm, tc_tkck, tc_illlist, tc_illcache, tc_decdim, tc_decw, tc_decmu;
     bool tc;
     // the tensor-core path for D > 128
-    size_t w_sd, w_kap, w_gd, w_phi, w_plo, w_tk, w_tkck, w_ckd, w_cref, w_illb, w_flags, w_yhi, w_ylo, w_logz, w_partial, w_llpart, w_illlist, w_muc, w_w2c, w_c2dc, w_statsc, w_top, w_logzx, w_compof, w_scra, w_scrw, w_scr, w_slotof, w_scrmask, w_n2, w_cand, w_candT, w_ctl, w_scre, w_slotcnt, w_heavyof, w_heavyslot, w_heavypart, w_scrahi, w_scrwhi, w_pairval, w_pairoff, w_pairbest;
+    size_t w_sd, w_kap, w_gd, w_phi, w_plo, w_tk, w_tkck, w_ckd, w_cref, w_illb, w_flags, w_yhi, w_ylo, w_logz, w_partial, w_llpart, w_illlist, w_muc, w_w2c, w_c2dc, w_statsc, w_top, w_logzx, w_compof, w_scra, w_scrw, w_scr, w_slotof, w_scrmask, w_n2, w_cand, w_candT, w_ctl, w_scre, w_slotcnt, w_heavyof, w_heavyslot, w_heavypart, w_scrahi, w_scrwhi, w_pairval, w_pairoff, w_pairbest, w_rec, w_reccnt, w_recthr;
     size_t w_partial_bytes;
     bool wide;
 };
@@ -89,7 +89,7 @@ ScratchLayout scratch_layout(int D, int K, bool planes) {
         L.tc_ylo = take(TC_YPLANE_BYTES);
     }
     L.w_sd = L.w_kap = L.w_gd = L.w_phi = L.w_plo = L.w_tk = L.w_tkck = L.w_ckd = L.w_cref = L.w_illb = L.w_flags = L.w_yhi = L.w_ylo = L.w_logz = L.w_partial = L.w_llpart = L.w_illlist = L.w_muc = L.w_w2c = L.w_c2dc = L.w_statsc = L.w_top = L.w_logzx = 0;
-    L.w_compof = L.w_scra = L.w_scrw = L.w_scr = L.w_slotof = L.w_scrmask = L.w_n2 = L.w_cand = L.w_candT = L.w_ctl = L.w_scre = L.w_slotcnt = L.w_heavyof = L.w_heavyslot = L.w_heavypart = L.w_scrahi = L.w_scrwhi = L.w_pairval = L.w_pairoff = L.w_pairbest = 0;
+    L.w_compof = L.w_scra = L.w_scrw = L.w_scr = L.w_slotof = L.w_scrmask = L.w_n2 = L.w_cand = L.w_candT = L.w_ctl = L.w_scre = L.w_slotcnt = L.w_heavyof = L.w_heavyslot = L.w_heavypart = L.w_scrahi = L.w_scrwhi = L.w_pairval = L.w_pairoff = L.w_pairbest = L.w_rec = L.w_reccnt = L.w_recthr = 0;
     L.w_partial_bytes = 0;
     L.wide = wide_supports(D, K) && planes;
     if (L.wide) {
@@ -126,6 +126,9 @@ ScratchLayout scratch_layout(int D, int K, bool planes) {
         L.w_pairval = take((size_t)WIDE_PAIR_VALS * 4);
         L.w_pairoff = take((size_t)WIDE_PIECE * 4);
         L.w_pairbest = take((size_t)WIDE_PIECE * 8);
+        L.w_rec = take((size_t)WIDE_PIECE * WIDE_REC * 4);
+        L.w_reccnt = take((size_t)WIDE_PIECE * 4);
+        L.w_recthr = take((size_t)WIDE_PIECE * 4);
         L.w_logz = take((size_t)WIDE_PIECE * 8);
         L.w_top = take((size_t)WIDE_PIECE * 2 * WIDE_MAX_TOP * 4);
         L.w_logzx = take((size_t)WIDE_PIECE * 8);
@@ -186,7 +189,8 @@ struct gmm_ctx {
     double wide_probe_limit = 0.0;   // automatic mode: "screen" while a sample of the points has at most this many marked pairs per
                                      // point (0: K / 300, or K / 24 below 128 points per component)
     bool wide_screen_all = false;    // the current step runs in "screen" mode
-    bool wide_pre = true;            // GMM_WIDE_PRE=0: no first pass for the screening threshold
+    bool wide_pre = false;           // GMM_WIDE_PRE=1: a first pass over the leading product for the screening threshold (instead
+                                     // of leaving the marks made against an immature threshold to the filter alone)
     bool wide_hi = true;             // GMM_WIDE_HI=0: the screening mode forms all three products for every component
     int wide_sparse = 1;             // GMM_WIDE_SPARSE: 0 = the listed components always go through the dense FP32 kernels,
                                      // 1 = pair by pair unless sweep 1 marks too many pairs, 2 = always pair by pair (tests)
@@ -290,6 +294,9 @@ struct gmm_ctx {
         b.pair_val = reinterpret_cast<float*>(scratch + lay.w_pairval);
         b.pair_off = reinterpret_cast<int*>(scratch + lay.w_pairoff);
         b.pair_best = reinterpret_cast<double*>(scratch + lay.w_pairbest);
+        b.rec = reinterpret_cast<unsigned*>(scratch + lay.w_rec);
+        b.rec_cnt = reinterpret_cast<int*>(scratch + lay.w_reccnt);
+        b.rec_thr = reinterpret_cast<float*>(scratch + lay.w_recthr);
         return b;
     }
 };
@@ -476,7 +483,8 @@ int prepare_and_choose(gmm_ctx* ctx, int64_t N, int D, int K, const float* pi, c
                 CU(launch_cand_clear_wide(ctx->stream, np, n_list, wb));
                 KL(launch_norm_wide(ctx->stream, Xprobe, np, D, wb));
                 KL(launch_transform_wide(ctx->stream, Xprobe, np, D, wb, &ctx->result()->status));
-                KL(launch_lse_wide(ctx->stream, np, D, K, fl[6], fl[4], n_list, wb, ctx->sms, &ctx->result()->status, 2, ctx->wide_hi ? fl[5] : -1, ctx->wide_pre));
+                KL(launch_lse_wide(ctx->stream, np, D, K, fl[6], fl[4], n_list, wb, ctx->sms, &ctx->result()->status, 2, ctx->wide_hi ? fl[5] : -1, ctx->wide_pre, true));
+                KL(launch_cand_filter_wide(ctx->stream, np, n_list, wb));
                 int marks = 0;
                 CU(cudaMemcpyAsync(&marks, wb.ctl, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
                 CU(cudaStreamSynchronize(ctx->stream));
@@ -582,7 +590,8 @@ int accumulate_points(gmm_ctx* ctx, int path, const float* X, int64_t n, int D, 
             CHECK(prof_begin(ctx));
             KL(launch_transform_wide(ctx->stream, Xs, cnt, D, wb, &ctx->result()->status));
             KL(launch_lse_wide(ctx->stream, cnt, D, K, Kg, screen ? n_listed : 0, n_ill, wb, ctx->sms, &ctx->result()->status, 2,
-                               (all && ctx->wide_hi) ? ctx->wide_n_first : -1, ctx->wide_pre));
+                               (all && ctx->wide_hi) ? ctx->wide_n_first : -1, ctx->wide_pre, true));
+            if (screen) KL(launch_cand_filter_wide(ctx->stream, cnt, n_ill, wb));
             if (ctx->wide_refine && !all) KL(launch_refine_wide(ctx->stream, Xs, cnt, D, K, mu, ctx->w2(), ctx->c2d(), wb));
             else CU(cudaMemcpyAsync(wb.logz_x, wb.logz, (size_t)cnt * 8, cudaMemcpyDeviceToDevice, ctx->stream));
             if (n_ill > 0) {
@@ -609,12 +618,12 @@ int accumulate_points(gmm_ctx* ctx, int path, const float* X, int64_t n, int D, 
                 }
                 if (n_a > 0) {
                     KL(launch_mstep_fp32(ctx->stream, Xs, cnt, D, n_a, wb.mu_c, wb.w2_c, wb.c2d_c, ctx->center(), wb.logz_x, ctx->partials(), plan_a, true, dense_if));
-                    KL(launch_reduce_partials(ctx->stream, D, n_a, plan_a.splits, ctx->partials(), ctx->center(), Nk_c, S1_c, S2_c, true));
+                    KL(launch_reduce_partials(ctx->stream, D, n_a, plan_a.splits, ctx->partials(), ctx->center(), Nk_c, S1_c, S2_c, true, dense_if));
                 }
                 if (n_b > 0) {
                     const size_t o = (size_t)n_a * D;
                     KL(launch_mstep_fp32(ctx->stream, Xs, cnt, D, n_b, wb.mu_c + o, wb.w2_c + o, wb.c2d_c + n_a, ctx->center(), wb.logz_x, ctx->partials(), plan_b, true, dense_if));
-                    KL(launch_reduce_partials(ctx->stream, D, n_b, plan_b.splits, ctx->partials(), ctx->center(), Nk_c + n_a, S1_c + o, S2_c + o, true));
+                    KL(launch_reduce_partials(ctx->stream, D, n_b, plan_b.splits, ctx->partials(), ctx->center(), Nk_c + n_a, S1_c + o, S2_c + o, true, dense_if));
                 }
                 if (screen) KL(launch_cand_count_wide(ctx->stream, wb));
             }

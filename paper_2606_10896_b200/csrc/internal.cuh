@@ -60,7 +60,7 @@ cudaError_t launch_topm_fp32(cudaStream_t s, const float* X, int64_t n, int D, i
 // each block being (N_k [K], sums of r (x - g) [K*D], sums of r (x - g)^2 [K*D]); float64 instead when
 // fp32_plan(D, K).wide.  g [D]: the centre launch_mstep_fp32 was given (NULL = 0); the shift back to S1, S2 is exact.
 cudaError_t launch_reduce_partials(cudaStream_t s, int D, int K, int splits, const float* partials, const float* g,
-                                   double* Nk, double* S1, double* S2, bool accumulate);
+                                   double* Nk, double* S1, double* S2, bool accumulate, const int* run_if = nullptr);
 // *ll (+)= sum of llpart[0..n) in a fixed order
 cudaError_t launch_reduce_ll(cudaStream_t s, const double* llpart, int64_t n, double* ll, bool accumulate);
 // counts (may be NULL): counts[0] += variance entries raised to the floor, counts[1] += components left unchanged

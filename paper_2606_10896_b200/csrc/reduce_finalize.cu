@@ -13,7 +13,8 @@ namespace {
 template <typename T>
 __global__ void reduce_partials_kernel(int D, int K, int splits, const T* __restrict__ partials,
                                        const float* __restrict__ g, double* __restrict__ Nk, double* __restrict__ S1,
-                                       double* __restrict__ S2, int accumulate) {
+                                       double* __restrict__ S2, int accumulate, const int* __restrict__ run_if) {
+    if (run_if && *run_if == 0) return;                  // (the kernel that fills the partials did not run either)
     const size_t KD = (size_t)K * D, per = (size_t)K + 2 * KD;
     const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (e >= per) return;
@@ -125,14 +126,14 @@ cudaError_t launch_finalize_isotropic(cudaStream_t s, int64_t N, int D, int K, c
 }
 
 cudaError_t launch_reduce_partials(cudaStream_t s, int D, int K, int splits, const float* partials, const float* g,
-                                   double* Nk, double* S1, double* S2, bool accumulate) {
+                                   double* Nk, double* S1, double* S2, bool accumulate, const int* run_if) {
     const size_t per = (size_t)K + 2 * (size_t)K * D;
     const unsigned blocks = (unsigned)((per + 255) / 256);
     if (fp32_plan(D, K).wide)
         reduce_partials_kernel<double><<<blocks, 256, 0, s>>>(D, K, splits, reinterpret_cast<const double*>(partials), g, Nk, S1, S2,
-                                                              accumulate ? 1 : 0);
+                                                              accumulate ? 1 : 0, run_if);
     else
-        reduce_partials_kernel<float><<<blocks, 256, 0, s>>>(D, K, splits, partials, g, Nk, S1, S2, accumulate ? 1 : 0);
+        reduce_partials_kernel<float><<<blocks, 256, 0, s>>>(D, K, splits, partials, g, Nk, S1, S2, accumulate ? 1 : 0, run_if);
     return cudaGetLastError();
 }
 

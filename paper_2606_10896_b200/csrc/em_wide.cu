@@ -38,6 +38,8 @@
 #include <cuda.h>
 #include <cuda_fp16.h>
 #include <math_constants.h>
+#include <cstdio>
+#include <cstdlib>
 #include <cstdlib>
 
 #define TC_WAIT_LIMIT_NS 2000000000ull
@@ -96,6 +98,7 @@ struct LseParams {
     unsigned* rec;       // NULL, or [n][WIDE_REC]: the marks' upper bounds, for the filter that follows
     int* rec_cnt;        // [n]
     float* rec_thr;      // [n] the point's final threshold
+    int dbg;
     int pre_pass;        // 1: before a tile's sweep proper, the groups from hi_group on are swept once for their lower bounds only
     int* ctl;
 };
@@ -138,12 +141,12 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
     __shared__ float top_s[128][2 * NTOP + 1];
     __shared__ float xm_s[256];
     // Per-component constants of the group at hand, one copy per warpgroup and two buffers (a warpgroup fills one while its
-    // slower warps may still read the other): (t, c, screening offset, screening slope), the allowance alone, the chunk masks.
+    // slower warps may still read the other): (t, c, screening offset, screening slope), the allowance alone, the slot, the chunk masks.
     // Read from global memory inside the loops over the accumulators they cost a trip to L2 per pair of components (the
     // shared-memory ring leaves almost no L1).
-    __shared__ int rcnt_s[128];                          // marks of the tile's points so far
     __shared__ float4 tab_s[2][2][128];
     __shared__ float tabe_s[2][2][128];
+    __shared__ int tabs_s[2][2][128];                    // (the slot of a listed component)
     __shared__ int tabm_s[2][2][4];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -160,7 +163,6 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
 
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L_BAR);
     auto BAR = [&](int i) { return smem_u32(&bars[i]); };
-    if (tid < 128) rcnt_s[tid] = 0;
     if (tid == 0) {
         abort_s = 0;
         drain_s = 0;
@@ -191,7 +193,7 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
         double ll_acc = 0.0;
         float2 n_tk = make_float2(0.f, 0.f), n_sc = make_float2(0.f, 0.f);
         float n_se = 0.f;
-        int n_mask = 0;
+        int n_mask = 0, n_slot = -1;
         auto table_load = [&](int g) {                       // this thread's component of the warpgroup's chunk of group g
             if (2 * g + grp < NC) {
                 const int col = (2 * g + grp) * 128 + pt;
@@ -199,6 +201,7 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
                 if (p.screen || NTOP > 2) n_sc = __ldg(p.scr + col);
                 if (p.screen) {
                     n_se = __ldg(p.scr_e + col);
+                    n_slot = __ldg(p.slot_of + col);
                     if (pt < 4) n_mask = __ldg(p.scr_mask + (col >> 5) + pt);
                 }
             }
@@ -206,6 +209,7 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
         auto table_store = [&](int tb) {
             tab_s[tb][grp][pt] = make_float4(n_tk.x, n_tk.y, n_sc.x, n_sc.y);
             tabe_s[tb][grp][pt] = n_se;
+            tabs_s[tb][grp][pt] = n_slot;
             if (pt < 4) tabm_s[tb][grp][pt] = n_mask;
         };
         for (int64_t i = 0; i < ntl; ++i) {
@@ -218,14 +222,16 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
             tl.init();
             // A pair that can matter: its bit in the map, and (for the filter that follows the sweep) its upper bound, rounded
             // up to the 19 bits that share a word with the slot.
-            auto mark = [&](float u, int col) {
-                const int sl = __ldg(p.slot_of + col);
-                if (sl < 0) return;
-                atomicOr(p.cand + row * p.cand_words + (sl >> 5), 1u << (sl & 31));
+            // (each warpgroup has its own half of the point's record)
+            int nrec = 0;
+            auto mark = [&](float u, int sl) {
+                if (sl < 0 || p.dbg == 3) return;
+                if (p.dbg != 1) atomicOr(p.cand + row * p.cand_words + (sl >> 5), 1u << (sl & 31));
                 ++nhit;
-                if (p.rec) {
-                    const int ri = atomicAdd(&rcnt_s[pt], 1);
-                    if (ri < WIDE_REC) p.rec[row * WIDE_REC + ri] = (__float_as_uint(u + fabsf(u) * 0.001953125f) & ~0x1FFFu) | (unsigned)sl;
+                if (p.rec && p.dbg != 2) {
+                    if (nrec < WIDE_REC / 2)
+                        p.rec[row * WIDE_REC + grp * (WIDE_REC / 2) + nrec] = (__float_as_uint(u + fabsf(u) * 0.001953125f) & ~0x1FFFu) | (unsigned)sl;
+                    ++nrec;
                 }
             };
             table_load(step_group(0));
@@ -311,8 +317,8 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
                                         thr_base = fmaxf(thr_base, fmaxf(u0 - 2.f * fmaf(sq.y, nrm, se.x), u1 - 2.f * fmaf(sq.w, nrm, se.y)));
                                         const float thr = thr_base - 40.f;
                                         if (ph == 0) continue;                          // (lower bounds only)
-                                        if (!(u0 < thr) && sq.x > -CUDART_INF_F) mark(u0, col0 + j);
-                                        if (!(u1 < thr) && sq.z > -CUDART_INF_F) mark(u1, col0 + j + 1);
+                                        if (!(u0 < thr) && sq.x > -CUDART_INF_F) mark(u0, tabs_s[tb][grp][sub * 32 + j]);
+                                        if (!(u1 < thr) && sq.z > -CUDART_INF_F) mark(u1, tabs_s[tb][grp][sub * 32 + j + 1]);
                                     }
                                 }
                                 continue;
@@ -373,7 +379,10 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
                 if (t + 1 < nsteps) table_store((int)(tcount & 1u));
             }
             // merge the two warpgroups' pairs; warpgroup 0 writes log2 Z and the two leading candidates
-            if (p.rec) xm_s[grp * 128 + pt] = thr_base;      // (each warpgroup's own slot; read after the barrier below)
+            if (p.rec) {
+                xm_s[grp * 128 + pt] = thr_base;             // (each warpgroup's own slot; read after the barrier below)
+                if (row < p.n) p.rec_cnt[2 * row + grp] = nrec;
+            }
             if (grp == 1) {
                 merge_s[pt] = make_float2(m_run, s_run);
 #pragma unroll
@@ -393,12 +402,8 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
 #pragma unroll
                     for (int j = 0; j < NTOP; ++j) { tp[j] = tl.a[j]; tp[NTOP + j] = __int_as_float(tl.i[j]); }
                     ll_acc += lz;
-                    if (p.rec) {
-                        p.rec_cnt[row] = rcnt_s[pt];
-                        p.rec_thr[row] = fmaxf(thr_base, xm_s[128 + pt]);
-                    }
+                    if (p.rec) p.rec_thr[row] = fmaxf(thr_base, xm_s[128 + pt]);
                 }
-                rcnt_s[pt] = 0;
             }
             if (nhit > 0) atomicAdd(p.ctl, nhit);
             named_bar_sync(2, 256);                          // merge_s is rewritten by the next tile
@@ -1253,7 +1258,7 @@ __global__ void __launch_bounds__(1024) wide_cref_kernel(int rows, const int* __
         const bool listed = slot_of[k] >= 0 && c >= 0 && isfinite(ckd[k]);
         // (hi_mode: the groups of 256 positions behind the first kind of listed components are screened by the leading
         // product alone, with the allowances that go with it)
-        const bool hi = hi_mode == 1 && k >= hi_start;
+        const bool hi = (hi_mode == 1 && k >= hi_start) || (hi_mode == 3 && k >= ((Kg + 255) & ~255));      // (3: every listed component)
         const float ea = listed ? (hi ? scra_hi[c] : scra[c]) : 0.f, ew = listed ? (hi ? scrw_hi[c] : scrw[c]) : 0.f;
         scr[k] = listed ? make_float2((float)fmin(ckd[k] - r + (double)ea, 3e38), ew)
                         : (in && c >= 0) ? (hi_mode == 2 ? make_float2(scra_hi[c], scrw_hi[c]) : make_float2(scra[c], scrw[c]))
@@ -1430,10 +1435,11 @@ __global__ void __launch_bounds__(256) wide_cand_filter_kernel(int64_t n, int wo
     const int64_t i = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (i >= n) return;
-    const int cnt = min(rec_cnt[i], WIDE_REC);
+    const int c0 = min(rec_cnt[2 * i], WIDE_REC / 2), c1 = min(rec_cnt[2 * i + 1], WIDE_REC / 2);     // the two halves of the record
     const float thr = rec_thr[i] - 40.f;
     int dropped = 0;
-    for (int r = lane; r < cnt; r += 32) {
+    for (int r = lane; r < WIDE_REC / 2 + c1; r += 32) {
+        if (r >= c0 && r < WIDE_REC / 2) continue;
         const unsigned v = rec[i * WIDE_REC + r];
         const int sl = (int)(v & 0x1FFFu);
         if (__uint_as_float(v & ~0x1FFFu) < thr) {           // (a NaN stays)
@@ -2364,6 +2370,7 @@ cudaError_t launch_lse_wide(cudaStream_t s, int64_t n, int D, int K, int Kg, int
     p.scr_e = wb.scr_e; p.scr_mask = wb.scr_mask; p.slot_of = wb.slot_of; p.n2 = wb.n2; p.cand = wb.cand;
     p.cand_words = (n_slots + 31) / 32; p.scr_group = Kgp / 256; p.ctl = wb.ctl;
     p.hi_group = 0x7fffffff; p.hi_end = 0x7fffffff; p.pre_pass = 0;
+    { const char* e = std::getenv("GMM_DBG"); p.dbg = e ? std::atoi(e) : 0; }
     p.rec = (record && screen && ntop == 2) ? wb.rec : nullptr; p.rec_cnt = wb.rec_cnt; p.rec_thr = wb.rec_thr;
     if (ntop == 2 && screen && hi_first_slots >= 0) {                                                      // the EM step's screening mode
         p.hi_group = (Kgp + hi_first_slots + 255) / 256;
@@ -2372,9 +2379,18 @@ cudaError_t launch_lse_wide(cudaStream_t s, int64_t n, int D, int K, int Kg, int
     if (ntop != 2 && hi_first_slots >= 0) { p.hi_group = 0; p.hi_end = Kgp / 256; }                         // the assignment's evaluated groups
     const int64_t ntiles = (n + WIDE_TILE - 1) / WIDE_TILE;
     const unsigned grid = (unsigned)(ntiles < num_sms ? ntiles : num_sms);
+    cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+    const bool timing = std::getenv("GMM_WIDE_TIMING") != nullptr;
+    if (timing) { cudaEventCreate(&ev0); cudaEventCreate(&ev1); cudaEventRecord(ev0, s); }
     if (ntop == 2) lse_wide_kernel<2><<<grid, WT_THREADS, L_SMEM, s>>>(p, tm_yhi, tm_ylo, tm_phi, tm_plo);
     else if (ntop == 6) lse_wide_kernel<6><<<grid, WT_THREADS, L_SMEM, s>>>(p, tm_yhi, tm_ylo, tm_phi, tm_plo);
     else lse_wide_kernel<WIDE_MAX_TOP><<<grid, WT_THREADS, L_SMEM, s>>>(p, tm_yhi, tm_ylo, tm_phi, tm_plo);
+    if (timing) {
+        cudaEventRecord(ev1, s); cudaEventSynchronize(ev1);
+        float ms = 0; cudaEventElapsedTime(&ms, ev0, ev1);
+        std::printf("lse_wide n=%lld %.3f ms\n", (long long)n, ms);
+        cudaEventDestroy(ev0); cudaEventDestroy(ev1);
+    }
     return cudaGetLastError();
 }
 

@@ -80,7 +80,8 @@ struct WideBuffers {
     int* heavy_slot;// [WIDE_HEAVY_SLOTS] the slot of each set of partial sums, -1 if unused
     double* heavy_part;    // [WIDE_HEAVY_SLOTS][WIDE_HEAVY_SEG][1 + 2 D] partial (N_k, S1, S2) of the split slots' segments
     unsigned* rec;     // [WIDE_PIECE][WIDE_REC] sweep 1's marks of a point: upper bound (rounded up to 19 bits) | slot (13 bits)
-    int* rec_cnt;      // [WIDE_PIECE] how many (may exceed WIDE_REC: the rest was not recorded)
+    int* rec_cnt;      // [WIDE_PIECE][2] how many in each half of a point's record (one half per softmax warpgroup; a count may
+                       // exceed the half's WIDE_REC / 2 entries: the rest was not recorded)
     float* rec_thr;    // [WIDE_PIECE] the point's final screening threshold (before the 2^-40 margin)
     float* pair_val;   // [WIDE_PAIR_VALS] exact log2 z of a piece's kept pairs relative to the point's best value, a point's
                        // marked pairs consecutive and in slot order (positions from a counter: ctl[4])

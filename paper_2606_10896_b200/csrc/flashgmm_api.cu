@@ -127,7 +127,7 @@ ScratchLayout scratch_layout(int D, int K, bool planes) {
         L.w_pairoff = take((size_t)WIDE_PIECE * 4);
         L.w_pairbest = take((size_t)WIDE_PIECE * 8);
         L.w_rec = take((size_t)WIDE_PIECE * WIDE_REC * 4);
-        L.w_reccnt = take((size_t)WIDE_PIECE * 4);
+        L.w_reccnt = take((size_t)WIDE_PIECE * 8);
         L.w_recthr = take((size_t)WIDE_PIECE * 4);
         L.w_logz = take((size_t)WIDE_PIECE * 8);
         L.w_top = take((size_t)WIDE_PIECE * 2 * WIDE_MAX_TOP * 4);
@@ -191,7 +191,9 @@ struct gmm_ctx {
     bool wide_screen_all = false;    // the current step runs in "screen" mode
     bool wide_pre = false;           // GMM_WIDE_PRE=1: a first pass over the leading product for the screening threshold (instead
                                      // of leaving the marks made against an immature threshold to the filter alone)
-    bool wide_hi = true;             // GMM_WIDE_HI=0: the screening mode forms all three products for every component
+    int wide_hi = 2;                 // GMM_WIDE_HI: which listed components the screening mode screens by the leading product alone:
+                                     // 0 = none (all three products for every component), 1 = those behind the first kind of the list
+                                     // (the components flagged by the rounding estimate keep all three products), 2 = all
     int wide_sparse = 1;             // GMM_WIDE_SPARSE: 0 = the listed components always go through the dense FP32 kernels,
                                      // 1 = pair by pair unless sweep 1 marks too many pairs, 2 = always pair by pair (tests)
     int tc_n_ill = 0;                // ill-conditioned components at the last result that was read back (picks the filter)
@@ -470,7 +472,7 @@ int prepare_and_choose(gmm_ctx* ctx, int64_t N, int D, int K, const float* pi, c
         // point: K / 24.
         const bool few_points = N < WIDE_AUTO_MIN_POINTS_PER_COMPONENT * K;
         if (ctx->wide_mode == 2 || (ctx->wide_mode == 0 && can_probe)) {
-            KL(launch_prepare_wide(ctx->stream, D, K, pi, mu, var, wb, limit, INFINITY, ctx->wide_hi ? 1 : 0));      // every component is listed
+            KL(launch_prepare_wide(ctx->stream, D, K, pi, mu, var, wb, limit, INFINITY, ctx->wide_hi == 2 ? 3 : ctx->wide_hi ? 1 : 0));      // every component is listed
             ctx->launches += 4;
             CU(cudaMemcpyAsync(fl, wb.flags, sizeof(fl), cudaMemcpyDeviceToHost, ctx->stream));
             CU(cudaStreamSynchronize(ctx->stream));
@@ -483,7 +485,7 @@ int prepare_and_choose(gmm_ctx* ctx, int64_t N, int D, int K, const float* pi, c
                 CU(launch_cand_clear_wide(ctx->stream, np, n_list, wb));
                 KL(launch_norm_wide(ctx->stream, Xprobe, np, D, wb));
                 KL(launch_transform_wide(ctx->stream, Xprobe, np, D, wb, &ctx->result()->status));
-                KL(launch_lse_wide(ctx->stream, np, D, K, fl[6], fl[4], n_list, wb, ctx->sms, &ctx->result()->status, 2, ctx->wide_hi ? fl[5] : -1, ctx->wide_pre, true));
+                KL(launch_lse_wide(ctx->stream, np, D, K, fl[6], fl[4], n_list, wb, ctx->sms, &ctx->result()->status, 2, ctx->wide_hi == 2 ? 0 : ctx->wide_hi ? fl[5] : -1, ctx->wide_pre, true));
                 KL(launch_cand_filter_wide(ctx->stream, np, n_list, wb));
                 int marks = 0;
                 CU(cudaMemcpyAsync(&marks, wb.ctl, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
@@ -491,6 +493,7 @@ int prepare_and_choose(gmm_ctx* ctx, int64_t N, int D, int K, const float* pi, c
                 const double auto_limit = (double)n_list / (few_points ? 24.0 : 300.0);
                 ok = (double)marks <= (ctx->wide_probe_limit > 0.0 ? ctx->wide_probe_limit : auto_limit) * (double)np;
             }
+            if (std::getenv("GMM_WIDE_TIMING")) std::printf("screen prepare: n_list %d n_ill %d first-kind slots %d Kg %d ok %d\n", n_list, fl[4], fl[5], fl[6], (int)ok);
             if (ok) {
                 ctx->wide_n_ill = fl[4];
                 ctx->wide_n_good = fl[6];
@@ -590,7 +593,7 @@ int accumulate_points(gmm_ctx* ctx, int path, const float* X, int64_t n, int D, 
             CHECK(prof_begin(ctx));
             KL(launch_transform_wide(ctx->stream, Xs, cnt, D, wb, &ctx->result()->status));
             KL(launch_lse_wide(ctx->stream, cnt, D, K, Kg, screen ? n_listed : 0, n_ill, wb, ctx->sms, &ctx->result()->status, 2,
-                               (all && ctx->wide_hi) ? ctx->wide_n_first : -1, ctx->wide_pre, true));
+                               !(all && ctx->wide_hi) ? -1 : ctx->wide_hi == 2 ? 0 : ctx->wide_n_first, ctx->wide_pre, true));
             if (screen) KL(launch_cand_filter_wide(ctx->stream, cnt, n_ill, wb));
             if (ctx->wide_refine && !all) KL(launch_refine_wide(ctx->stream, Xs, cnt, D, K, mu, ctx->w2(), ctx->c2d(), wb));
             else CU(cudaMemcpyAsync(wb.logz_x, wb.logz, (size_t)cnt * 8, cudaMemcpyDeviceToDevice, ctx->stream));
@@ -744,7 +747,7 @@ int gmm_create(gmm_ctx** out, int device, void* cuda_stream) {
     if (const char* e = std::getenv("GMM_WIDE_MIN_POINTS")) ctx->wide_min_points = std::atof(e);
     if (const char* e = std::getenv("GMM_WIDE_REFINE")) ctx->wide_refine = std::atoi(e) != 0;
     if (const char* e = std::getenv("GMM_WIDE_SPARSE")) ctx->wide_sparse = std::atoi(e);
-    if (const char* e = std::getenv("GMM_WIDE_HI")) ctx->wide_hi = std::atoi(e) != 0;
+    if (const char* e = std::getenv("GMM_WIDE_HI")) ctx->wide_hi = std::atoi(e);
     if (const char* e = std::getenv("GMM_WIDE_PRE")) ctx->wide_pre = std::atoi(e) != 0;
     if (const char* e = std::getenv("GMM_WIDE_MODE")) ctx->wide_mode = !std::strcmp(e, "sweeps") ? 1 : !std::strcmp(e, "screen") ? 2 : 0;
     if (const char* e = std::getenv("GMM_WIDE_PROBE_LIMIT")) ctx->wide_probe_limit = std::atof(e);
@@ -1060,7 +1063,7 @@ int assign_topm_impl(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, cons
             // (indices only: the sweep forms the leading fp16 product alone for the evaluated components - a third of the tensor
             // work - and ranks by correspondingly wider bounds; with responsibilities asked for, the approximate log Z has to
             // be good and all three products are formed)
-            const bool hi = index_only && ctx->wide_hi;
+            const bool hi = index_only && ctx->wide_hi != 0;
             KL(launch_prepare_wide(ctx->stream, D, K, pi, mu, var, wb, limit, 0.f, hi ? 2 : 0));
             ctx->launches += 4;
             int fl[8];

@@ -99,6 +99,7 @@ struct LseParams {
     int* rec_cnt;        // [n]
     float* rec_thr;      // [n] the point's final threshold
     int dbg;
+    int g0;              // the sweep starts at this group (the "screen" mode: behind the unlisted components, which have no weight)
     int pre_pass;        // 1: before a tile's sweep proper, the groups from hi_group on are swept once for their lower bounds only
     int* ctl;
 };
@@ -157,8 +158,8 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
     // A tile's steps, the same for every role: with pre_pass the groups from hi_group on once for their lower bounds (so that
     // the threshold is final before anything is marked), then every group.
     const int npre = (p.pre_pass && p.hi_group < NG) ? NG - p.hi_group : 0;
-    const int nsteps = npre + NG;
-    auto step_group = [&](int t) { return t < npre ? p.hi_group + t : t - npre; };
+    const int nsteps = npre + NG - p.g0;
+    auto step_group = [&](int t) { return t < npre ? p.hi_group + t : p.g0 + t - npre; };
     auto leading_only = [&](int g) { return g >= p.hi_group && g < p.hi_end; };
 
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L_BAR);
@@ -2341,7 +2342,7 @@ cudaError_t launch_transform_wide(cudaStream_t s, const float* X, int64_t n, int
 }
 
 cudaError_t launch_lse_wide(cudaStream_t s, int64_t n, int D, int K, int Kg, int n_listed, int n_slots, const WideBuffers& wb,
-                            int num_sms, int* status, int ntop, int hi_first_slots, bool pre_pass, bool record) {
+                            int num_sms, int* status, int ntop, int hi_first_slots, bool pre_pass, bool record, bool listed_only) {
     if (n < 1 || n > WIDE_PIECE || Kg < 0 || Kg > K || (Kg < 1 && n_listed < 1)) return cudaErrorInvalidValue;
     const WidePlan pl = wide_plan(D, K, num_sms);
     const int64_t rp = rows_padded_of(n);
@@ -2371,6 +2372,7 @@ cudaError_t launch_lse_wide(cudaStream_t s, int64_t n, int D, int K, int Kg, int
     p.cand_words = (n_slots + 31) / 32; p.scr_group = Kgp / 256; p.ctl = wb.ctl;
     p.hi_group = 0x7fffffff; p.hi_end = 0x7fffffff; p.pre_pass = 0;
     { const char* e = std::getenv("GMM_DBG"); p.dbg = e ? std::atoi(e) : 0; }
+    p.g0 = (listed_only && screen && ntop == 2) ? Kgp / 256 : 0;
     p.rec = (record && screen && ntop == 2) ? wb.rec : nullptr; p.rec_cnt = wb.rec_cnt; p.rec_thr = wb.rec_thr;
     if (ntop == 2 && screen && hi_first_slots >= 0) {                                                      // the EM step's screening mode
         p.hi_group = (Kgp + hi_first_slots + 255) / 256;

@@ -129,7 +129,9 @@ cudaError_t launch_cand_count_wide(cudaStream_t s, const WideBuffers& wb);
 // 256 positions behind them are screened by the leading product alone.
 cudaError_t launch_lse_wide(cudaStream_t s, int64_t n, int D, int K, int Kg, int n_listed, int n_slots, const WideBuffers& wb,
                             int num_sms, int* status, int ntop = 2, int hi_first_slots = -1, bool pre_pass = false,
-                            bool record = false);
+                            bool record = false, bool listed_only = false);
+// listed_only: the sweep leaves out the groups of the unlisted components (the caller knows that none of them has a weight;
+// wb.logz is then -inf for every point).
 // record (screening, ntop = 2): every mark's upper bound goes to wb.rec and the point's final threshold to wb.rec_thr, for
 // launch_cand_filter_wide.
 // pre_pass (with hi_first_slots >= 0): every tile first sweeps those groups once for the largest lower bound alone, so that

@@ -195,6 +195,7 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
         float2 n_tk = make_float2(0.f, 0.f), n_sc = make_float2(0.f, 0.f);
         float n_se = 0.f;
         int n_mask = 0, n_slot = -1;
+        int nhit = 0;                                        // pairs this thread has marked (all tiles)
         auto table_load = [&](int g) {                       // this thread's component of the warpgroup's chunk of group g
             if (2 * g + grp < NC) {
                 const int col = (2 * g + grp) * 128 + pt;
@@ -218,7 +219,6 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
             float m_run = -1e30f, s_run = 0.f;               // finite start: blocks of -inf logits must not make NaN
             const float nrm = ((p.screen || NTOP > 2) && row < p.n) ? __ldg(p.n2 + row) : 0.f;
             float thr_base = -1e30f;
-            int nhit = 0;
             WideTop<NTOP> tl;                                // the largest logits of this thread's chunks, and where
             tl.init();
             // A pair that can matter: its bit in the map, and (for the filter that follows the sweep) its upper bound, rounded
@@ -406,9 +406,13 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
                     if (p.rec) p.rec_thr[row] = fmaxf(thr_base, xm_s[128 + pt]);
                 }
             }
-            if (nhit > 0) atomicAdd(p.ctl, nhit);
             named_bar_sync(2, 256);                          // merge_s is rewritten by the next tile
         }
+        // (one addition per warp: an addition per thread and tile, all to one address, kept an L2 slice busy for a third
+        // of the sweep's time)
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) nhit += __shfl_xor_sync(0xffffffffu, nhit, o);
+        if (lane == 0 && nhit > 0) atomicAdd(p.ctl, nhit);
         if (grp == 0) ll_s[pt] = ll_acc;
         named_bar_sync(1, 256);
         if (tid == 0 && p.llpart) {
@@ -1433,13 +1437,14 @@ __global__ void __launch_bounds__(256) wide_norm_kernel(const float* __restrict_
 __global__ void __launch_bounds__(256) wide_cand_filter_kernel(int64_t n, int words, unsigned* __restrict__ cand,
                                                                const unsigned* __restrict__ rec, const int* __restrict__ rec_cnt,
                                                                const float* __restrict__ rec_thr, int* __restrict__ ctl) {
+    __shared__ int drop_s[8];
     const int64_t i = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
-    if (i >= n) return;
-    const int c0 = min(rec_cnt[2 * i], WIDE_REC / 2), c1 = min(rec_cnt[2 * i + 1], WIDE_REC / 2);     // the two halves of the record
-    const float thr = rec_thr[i] - 40.f;
+    const bool in = i < n;
+    const int c0 = in ? min(rec_cnt[2 * i], WIDE_REC / 2) : 0, c1 = in ? min(rec_cnt[2 * i + 1], WIDE_REC / 2) : 0;     // the two halves of the record
+    const float thr = in ? rec_thr[i] - 40.f : 0.f;
     int dropped = 0;
-    for (int r = lane; r < WIDE_REC / 2 + c1; r += 32) {
+    for (int r = lane; in && r < WIDE_REC / 2 + c1; r += 32) {
         if (r >= c0 && r < WIDE_REC / 2) continue;
         const unsigned v = rec[i * WIDE_REC + r];
         const int sl = (int)(v & 0x1FFFu);
@@ -1450,7 +1455,13 @@ __global__ void __launch_bounds__(256) wide_cand_filter_kernel(int64_t n, int wo
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) dropped += __shfl_xor_sync(0xffffffffu, dropped, o);
-    if (lane == 0 && dropped > 0) atomicSub(ctl, dropped);
+    if (lane == 0) drop_s[threadIdx.x >> 5] = dropped;
+    __syncthreads();
+    if (threadIdx.x == 0) {                                  // (one subtraction per block: they all go to one address)
+        int t = 0;
+        for (int w = 0; w < 8; ++w) t += drop_s[w];
+        if (t > 0) atomicSub(ctl, t);
+    }
 }
 
 __global__ void wide_cand_gate_kernel(int* __restrict__ ctl, long long max_pairs) {
@@ -1461,10 +1472,21 @@ __global__ void wide_cand_gate_kernel(int* __restrict__ ctl, long long max_pairs
 
 // Per-step totals for diagnostics: flags[1] += pairs marked, flags[3] += pairs kept, flags[7] += 1 for a piece that went
 // through the dense kernels (saturating).
-__global__ void wide_cand_count_kernel(const int* __restrict__ ctl, int* __restrict__ flags) {
-    auto add = [](int a, int b) { const long long t = (long long)a + (long long)b; return t > 2147483647LL ? 2147483647 : (int)t; };
+__global__ void __launch_bounds__(256) wide_cand_count_kernel(const int* __restrict__ ctl, int* __restrict__ flags,
+                                                              const int* __restrict__ slot_cnt, int n_slots) {
+    __shared__ long long red[256];
+    long long k = 0;                                         // pairs kept: the slots' counts
+    for (int j = threadIdx.x; j < n_slots; j += 256) k += slot_cnt[j];
+    red[threadIdx.x] = k;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) {
+        if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o];
+        __syncthreads();
+    }
+    if (threadIdx.x != 0) return;
+    auto add = [](int a, long long b) { const long long t = (long long)a + b; return t > 2147483647LL ? 2147483647 : (int)t; };
     flags[1] = add(flags[1], ctl[0]);
-    flags[3] = add(flags[3], ctl[1] ? 0 : ctl[3]);
+    flags[3] = add(flags[3], ctl[1] ? 0 : red[0]);
     flags[7] = add(flags[7], ctl[1] ? 1 : 0);
 }
 
@@ -1517,20 +1539,39 @@ __global__ void __launch_bounds__(256, 4) wide_cand_lse_kernel(const float* __re
     if (ctl[1] != 0) return;
     __shared__ double lbuf[8][CAND_KEEP];
     __shared__ unsigned short slist[8][CAND_LIST];
+    __shared__ int tot_s[8];
+    __shared__ int base_s;
     const int64_t i = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    if (i >= n) return;
     unsigned bits[CAND_WORDS_PER_LANE];
-    unsigned any = 0u;
+    int nmarked = 0;
 #pragma unroll
     for (int q = 0; q < CAND_WORDS_PER_LANE; ++q) {
-        bits[q] = (lane + 32 * q < words) ? cand[i * words + lane + 32 * q] : 0u;
-        any |= bits[q];
+        bits[q] = (i < n && lane + 32 * q < words) ? cand[i * words + lane + 32 * q] : 0u;
+        nmarked += __popc(bits[q]);
     }
-    if (!__any_sync(0xffffffffu, any != 0u)) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) nmarked += __shfl_xor_sync(0xffffffffu, nmarked, o);
+    // Room for the exact values of the block's pairs (the statistics kernel reads them back instead of evaluating its pairs
+    // again): one request per block - they all go to one counter.  Where the room starts depends on timing, what is stored
+    // there does not.  No room left: ctl[5] tells the statistics kernel to evaluate every pair of the piece itself.
+    if (lane == 0) tot_s[w] = nmarked;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int t = 0;
+        for (int j = 0; j < 8; ++j) t += tot_s[j];
+        int b = t > 0 ? atomicAdd(ctl + 4, t) : 0;
+        if (b < 0 || b > WIDE_PAIR_VALS - t) { b = -1; ctl[5] = 1; }
+        base_s = b;
+    }
+    __syncthreads();
+    if (i >= n) return;
+    if (nmarked == 0) {
         if (lane == 0) out[i] = -CUDART_INF;
         return;
     }
+    int off = base_s;
+    for (int j = 0; j < w; ++j) off += (off >= 0) ? tot_s[j] : 0;
     const float* xr = X + i * D;
     auto word_at = [&](int wi) {
         unsigned v = bits[0];
@@ -1665,15 +1706,6 @@ __global__ void __launch_bounds__(256, 4) wide_cand_lse_kernel(const float* __re
     }
     __syncwarp();
     const bool listed = total <= CAND_LIST;                   // (else: the row is scanned word by word, as a fallback)
-    // Room for the exact values of the point's pairs (the statistics kernel reads them back instead of evaluating its pairs
-    // again).  Where the room starts depends on timing, what is stored there does not.  No room left: ctl[5] tells the
-    // statistics kernel to evaluate every pair of the piece itself.
-    int off = -1;
-    if (lane == 0) {
-        off = atomicAdd(ctl + 4, total);
-        if (off < 0 || off > WIDE_PAIR_VALS - total) { off = -1; ctl[5] = 1; }
-    }
-    off = __shfl_sync(0xffffffffu, off, 0);
     double best = logz[i];
     int idx = 0;
     {
@@ -1749,7 +1781,6 @@ __global__ void __launch_bounds__(256, 4) wide_cand_lse_kernel(const float* __re
     }
     if (lane == 0) {
         out[i] = kept ? m + log2(ssum) : -CUDART_INF;
-        if (kept) atomicAdd(ctl + 3, kept);
         pair_off[i] = off;
         pair_best[i] = best;
     }
@@ -2284,8 +2315,8 @@ cudaError_t launch_cand_gate_wide(cudaStream_t s, const WideBuffers& wb, long lo
     return cudaGetLastError();
 }
 
-cudaError_t launch_cand_count_wide(cudaStream_t s, const WideBuffers& wb) {
-    wide_cand_count_kernel<<<1, 1, 0, s>>>(wb.ctl, wb.flags);
+cudaError_t launch_cand_count_wide(cudaStream_t s, int n_slots, const WideBuffers& wb) {
+    wide_cand_count_kernel<<<1, 256, 0, s>>>(wb.ctl, wb.flags, wb.slot_cnt, n_slots);
     return cudaGetLastError();
 }
 

@@ -117,9 +117,9 @@ cudaError_t launch_merge_ll_wide(cudaStream_t s, int64_t n, const WideBuffers& w
 // stats rows of the listed components += wb.stats_c.
 cudaError_t launch_ill_scatter_wide(cudaStream_t s, int D, int K, int n_ill, const WideBuffers& wb, double* Nk, double* S1,
                                     double* S2);
-// wb.flags[1] += wb.ctl[0] (pairs marked), wb.flags[3] += wb.ctl[3] (pairs kept), wb.flags[7] += 1 if the piece went through
+// wb.flags[1] += wb.ctl[0] (pairs marked), wb.flags[3] += the sum of wb.slot_cnt (pairs kept), wb.flags[7] += 1 if the piece went through
 // the dense kernels: totals of a step, for diagnostics.
-cudaError_t launch_cand_count_wide(cudaStream_t s, const WideBuffers& wb);
+cudaError_t launch_cand_count_wide(cudaStream_t s, int n_slots, const WideBuffers& wb);
 // First sweep over the n points whose planes were written: log2 Z per point over the Kg evaluated components -> wb.logz.
 // n_listed > 0 (listed components, n_slots slots of the list): the sweep also marks in wb.cand every pair of a point and a
 // listed component whose approximate log2 z, raised by its error bound, comes within 2^-40 of the point's maximum, and

@@ -628,7 +628,7 @@ int accumulate_points(gmm_ctx* ctx, int path, const float* X, int64_t n, int D, 
                     KL(launch_mstep_fp32(ctx->stream, Xs, cnt, D, n_b, wb.mu_c + o, wb.w2_c + o, wb.c2d_c + n_a, ctx->center(), wb.logz_x, ctx->partials(), plan_b, true, dense_if));
                     KL(launch_reduce_partials(ctx->stream, D, n_b, plan_b.splits, ctx->partials(), ctx->center(), Nk_c + n_a, S1_c + o, S2_c + o, true, dense_if));
                 }
-                if (screen) KL(launch_cand_count_wide(ctx->stream, wb));
+                if (screen) KL(launch_cand_count_wide(ctx->stream, n_ill, wb));
             }
             CHECK(prof_end(ctx));                             // (the bracket holds every kernel of the piece)
         }

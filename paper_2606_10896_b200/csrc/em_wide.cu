@@ -1529,7 +1529,7 @@ constexpr int CAND_WORDS_PER_LANE = (WIDE_CAND_WORDS + 31) / 32;
 constexpr int CAND_KEEP = 256;          // exact values of a point's first pairs kept between the two rounds
 constexpr int CAND_LIST = 256;          // marked slots of a point listed in shared memory (more: the row is scanned instead)
 constexpr int CAND_G = 4;               // marked pairs of a point taken together (their loads overlap)
-__global__ void __launch_bounds__(256, 4) wide_cand_lse_kernel(const float* __restrict__ X, int64_t n, int D, int words,
+__global__ void __launch_bounds__(256, 3) wide_cand_lse_kernel(const float* __restrict__ X, int64_t n, int D, int words,
                                                             const unsigned* __restrict__ cand, unsigned* __restrict__ candT,
                                                             const float* __restrict__ mu_c, const float* __restrict__ w2_c,
                                                             const double* __restrict__ c2d_c, const double* __restrict__ logz,
@@ -1600,25 +1600,35 @@ __global__ void __launch_bounds__(256, 4) wide_cand_lse_kernel(const float* __re
         const float room = (stop > -CUDART_INF) ? (float)fmin(fmax(c - stop + 1.0, -3e38), 3e38) : CUDART_INF_F;
         double q = 0.0;
         float run = 0.f;
+        // (four chunks of 128 dimensions at a time: their loads are in flight together, and the running total is looked at
+        // after each four - with a final threshold nearly every pair that gets here is kept, and a look after every chunk
+        // or two made the evaluation a chain of five trips to L2)
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            if (128 * j < D) {                               // warp-uniform
-                float part = 0.f;
-                if (128 * j + 4 * lane < D) {
-                    const float4 m4 = __ldg(mr + 32 * j), w4 = __ldg(wr + 32 * j);
-                    float dd = xq[j].x - m4.x;  part = fmaf(dd * dd, w4.x, part);
-                    dd = xq[j].y - m4.y;        part = fmaf(dd * dd, w4.y, part);
-                    dd = xq[j].z - m4.z;        part = fmaf(dd * dd, w4.z, part);
-                    dd = xq[j].w - m4.w;        part = fmaf(dd * dd, w4.w, part);
-                }
-                q += (double)part;
-                run += part;
-                if (j == 0 || (j & 1) == 0) {                // after 128 dimensions, then after every 256
-                    float tot = run;
+        for (int h = 0; h < 2; ++h) {
+            if (512 * h < D) {                               // warp-uniform
+                float4 m4[4], w4[4];
 #pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, o);
-                    if (tot > room) return -CUDART_INF;
+                for (int jj = 0; jj < 4; ++jj) {
+                    const int j = 4 * h + jj;
+                    const bool in = 128 * j + 4 * lane < D;
+                    m4[jj] = in ? __ldg(mr + 32 * j) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    w4[jj] = in ? __ldg(wr + 32 * j) : make_float4(0.f, 0.f, 0.f, 0.f);
                 }
+#pragma unroll
+                for (int jj = 0; jj < 4; ++jj) {
+                    const int j = 4 * h + jj;
+                    float part = 0.f;
+                    float dd = xq[j].x - m4[jj].x;  part = fmaf(dd * dd, w4[jj].x, part);
+                    dd = xq[j].y - m4[jj].y;        part = fmaf(dd * dd, w4[jj].y, part);
+                    dd = xq[j].z - m4[jj].z;        part = fmaf(dd * dd, w4[jj].z, part);
+                    dd = xq[j].w - m4[jj].w;        part = fmaf(dd * dd, w4[jj].w, part);
+                    q += (double)part;
+                    run += part;
+                }
+                float tot = run;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, o);
+                if (tot > room) return -CUDART_INF;
             }
         }
 #pragma unroll

@@ -187,7 +187,7 @@ struct gmm_ctx {
     int wide_mode = 0;               // GMM_WIDE_MODE: 0 = automatic, 1 = "sweeps" (two tensor sweeps, few components exact),
                                      // 2 = "screen" (one tensor sweep screens every pair, every component evaluated exactly)
     double wide_probe_limit = 0.0;   // automatic mode: "screen" while a sample of the points has at most this many marked pairs per
-                                     // point (0: K / 300, or K / 24 below 128 points per component)
+                                     // point (0: K / 200, or K / 16 below 128 points per component)
     bool wide_screen_all = false;    // the current step runs in "screen" mode
     bool wide_pre = false;           // GMM_WIDE_PRE=1: a first pass over the leading product for the screening threshold (instead
                                      // of leaving the marks made against an immature threshold to the filter alone)
@@ -462,14 +462,13 @@ int prepare_and_choose(gmm_ctx* ctx, int64_t N, int D, int K, const float* pi, c
         int fl[8];
         const bool can_probe = Xprobe != nullptr && n_probe >= 1;
         // Automatic choice, step by step: the screening sweep is tried on the first 8192 rows, and "screen" is taken if it marks
-        // few enough pairs per point.  With the threshold final before anything is marked, nearly every marked pair is kept,
-        // and a kept pair costs 4-7 ns at D = 768 (exact evaluation plus its statistics: measured 43-76 ms per 10 million
-        // points and pair per point).  What "screen" saves is the second tensor sweep, whose cost per point grows with K D
-        // like the pair's does with D: from 128 points per component on the limit is K / 400 marked pairs per point
-        // (config 5: 10; its iterations from a data-row initialisation mark 9, 30, 11, 4.6, 3.3 and take 0.88, 2.05, 0.96,
-        // 0.72, 0.68 s in "screen" against 1.24, 1.28, 1.04, 1.06, 1.06 s in "sweeps").  Below 128 points per component
-        // "sweeps" is no alternative (it would list most components as light) and the FP32 kernels cost K D / 2 ns per
-        // point: K / 24.
+        // few enough pairs per point.  With the marks filtered against the final threshold nearly every marked pair is kept,
+        // and a kept pair costs 3.6 ns at D = 768 (exact evaluation plus its statistics); the mode's fixed part is 16 ns per
+        // point at config 5's shape.  What "screen" saves is the second tensor sweep and the two low-order products of the
+        // first (config 5: 104 against 16 ns per point), whose cost per point grows with K D like the pair's does with D:
+        // from 128 points per component on the limit is K / 200 marked pairs per point (config 5: 20; its iterations from a
+        // data-row initialisation mark 9, 30, 11, 4.5, 3.3, 2.9).  Below 128 points per component "sweeps" is no alternative
+        // (it would list most components as light) and the FP32 kernels cost K D / 2 ns per point: K / 16.
         const bool few_points = N < WIDE_AUTO_MIN_POINTS_PER_COMPONENT * K;
         if (ctx->wide_mode == 2 || (ctx->wide_mode == 0 && can_probe)) {
             KL(launch_prepare_wide(ctx->stream, D, K, pi, mu, var, wb, limit, INFINITY, ctx->wide_hi == 2 ? 3 : ctx->wide_hi ? 1 : 0));      // every component is listed
@@ -490,7 +489,7 @@ int prepare_and_choose(gmm_ctx* ctx, int64_t N, int D, int K, const float* pi, c
                 int marks = 0;
                 CU(cudaMemcpyAsync(&marks, wb.ctl, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
                 CU(cudaStreamSynchronize(ctx->stream));
-                const double auto_limit = (double)n_list / (few_points ? 24.0 : 300.0);
+                const double auto_limit = (double)n_list / (few_points ? 16.0 : 200.0);
                 ok = (double)marks <= (ctx->wide_probe_limit > 0.0 ? ctx->wide_probe_limit : auto_limit) * (double)np;
             }
             if (std::getenv("GMM_WIDE_TIMING")) std::printf("screen prepare: n_list %d n_ill %d first-kind slots %d Kg %d ok %d\n", n_list, fl[4], fl[5], fl[6], (int)ok);
@@ -602,7 +601,7 @@ int accumulate_points(gmm_ctx* ctx, int path, const float* X, int64_t n, int D, 
                     // more than one pair in 64 marked (or the pair-by-pair route switched off): the dense kernels are cheaper
                     // ("screen" mode: the dense alternative evaluates every component, so the pair route pays for longer)
                     const long long max_pairs = ctx->wide_sparse >= 2 ? ((long long)1 << 62)
-                                              : all ? (long long)cnt * n_ill / 24 : (long long)cnt * n_ill / 64;
+                                              : all ? (long long)cnt * n_ill / 16 : (long long)cnt * n_ill / 64;
                     KL(launch_cand_gate_wide(ctx->stream, wb, max_pairs));
                     KL(launch_cand_lse_wide(ctx->stream, Xs, cnt, D, n_ill, wb, ctx->logZ2()));
                 }

@@ -920,11 +920,13 @@ __global__ void __launch_bounds__(256) wide_transform_kernel(const float* __rest
         }
         const size_t o = ((size_t)(ks >> 2) * rows_padded + row) * 128 + (ks & 3) * 32;      // [atom][row][128 bytes]
         uint4* oh = reinterpret_cast<uint4*>(yhi + o);
-        uint4* ol = reinterpret_cast<uint4*>(ylo + o);
         oh[0] = make_uint4(xh[0], xh[1], xh[2], xh[3]);
         oh[1] = make_uint4(qh[0], qh[1], qh[2], qh[3]);
-        ol[0] = make_uint4(xl[0], xl[1], xl[2], xl[3]);
-        ol[1] = make_uint4(ql[0], ql[1], ql[2], ql[3]);
+        if (ylo) {                                           // (NULL: the sweep that follows forms leading products only)
+            uint4* ol = reinterpret_cast<uint4*>(ylo + o);
+            ol[0] = make_uint4(xl[0], xl[1], xl[2], xl[3]);
+            ol[1] = make_uint4(ql[0], ql[1], ql[2], ql[3]);
+        }
     }
     if (bad) atomicOr(status, ST_BAD_X);
 }
@@ -2371,14 +2373,14 @@ cudaError_t launch_assign_refine_wide(cudaStream_t s, const float* X, int64_t n,
     return cudaGetLastError();
 }
 
-cudaError_t launch_transform_wide(cudaStream_t s, const float* X, int64_t n, int D, const WideBuffers& wb, int* status) {
+cudaError_t launch_transform_wide(cudaStream_t s, const float* X, int64_t n, int D, const WideBuffers& wb, int* status, bool hi_only) {
     if (n < 1 || n > WIDE_PIECE) return cudaErrorInvalidValue;
     const WidePlan pl = wide_plan(D, 1, 148);
     const int64_t rp = rows_padded_of(n);
     const int64_t units = rp * (pl.Dpad >> 3);
     int64_t blocks = (units + 255) / 256;
     if (blocks > 148 * 16) blocks = 148 * 16;
-    wide_transform_kernel<<<(unsigned)blocks, 256, 0, s>>>(X, n, rp, D, pl.Dpad, wb.sd, wb.kap, wb.gd, wb.y_hi, wb.y_lo, status);
+    wide_transform_kernel<<<(unsigned)blocks, 256, 0, s>>>(X, n, rp, D, pl.Dpad, wb.sd, wb.kap, wb.gd, wb.y_hi, hi_only ? nullptr : wb.y_lo, status);
     return cudaGetLastError();
 }
 

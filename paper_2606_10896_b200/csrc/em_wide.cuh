@@ -103,7 +103,8 @@ cudaError_t launch_prepare_wide(cudaStream_t s, int D, int K, const float* pi, c
 // hi_mode 2 (the assignment): the evaluated components get them; launch_lse_wide (ntop > 2) is given hi_first_slots = 0
 // and launch_assign_refine_wide hi = true.
 // n <= WIDE_PIECE points: X -> the fp16 planes of Y (rows up to the next multiple of 256 are written as zeros).
-cudaError_t launch_transform_wide(cudaStream_t s, const float* X, int64_t n, int D, const WideBuffers& wb, int* status);
+cudaError_t launch_transform_wide(cudaStream_t s, const float* X, int64_t n, int D, const WideBuffers& wb, int* status,
+                                  bool hi_only = false);       // hi_only: the lo plane is not written (a sweep of leading products follows)
 // The listed components' rows of the FP32 path's derived parameters packed into wb.mu_c / w2_c / c2d_c.
 cudaError_t launch_ill_gather_wide(cudaStream_t s, int D, int n_ill, const WideBuffers& wb, const float* mu, const float* w2,
                                    const double* c2d);

@@ -483,7 +483,7 @@ int prepare_and_choose(gmm_ctx* ctx, int64_t N, int D, int K, const float* pi, c
                 const int64_t np = n_probe < 8192 ? n_probe : 8192;
                 CU(launch_cand_clear_wide(ctx->stream, np, n_list, wb));
                 KL(launch_norm_wide(ctx->stream, Xprobe, np, D, wb));
-                KL(launch_transform_wide(ctx->stream, Xprobe, np, D, wb, &ctx->result()->status));
+                KL(launch_transform_wide(ctx->stream, Xprobe, np, D, wb, &ctx->result()->status, ctx->wide_hi == 2));
                 KL(launch_lse_wide(ctx->stream, np, D, K, fl[6], fl[4], n_list, wb, ctx->sms, &ctx->result()->status, 2, ctx->wide_hi == 2 ? 0 : ctx->wide_hi ? fl[5] : -1, ctx->wide_pre, true, true));
                 KL(launch_cand_filter_wide(ctx->stream, np, n_list, wb));
                 int marks = 0;
@@ -590,7 +590,7 @@ int accumulate_points(gmm_ctx* ctx, int path, const float* X, int64_t n, int D, 
                 KL(launch_norm_wide(ctx->stream, Xs, cnt, D, wb));
             }
             CHECK(prof_begin(ctx));
-            KL(launch_transform_wide(ctx->stream, Xs, cnt, D, wb, &ctx->result()->status));
+            KL(launch_transform_wide(ctx->stream, Xs, cnt, D, wb, &ctx->result()->status, all && ctx->wide_hi == 2));
             KL(launch_lse_wide(ctx->stream, cnt, D, K, Kg, screen ? n_listed : 0, n_ill, wb, ctx->sms, &ctx->result()->status, 2,
                                !(all && ctx->wide_hi) ? -1 : ctx->wide_hi == 2 ? 0 : ctx->wide_n_first, ctx->wide_pre, true, all));
             if (screen) KL(launch_cand_filter_wide(ctx->stream, cnt, n_ill, wb));

@@ -936,15 +936,25 @@ __device__ __forceinline__ void tc_store_unit(const float (&x)[8], bool valid, c
                                               unsigned char* __restrict__ yhi, unsigned char* __restrict__ ylo) {
     const int64_t row = u >> 4;
     const int ks = (int)(u & 15), d0 = ks * 8;
+    // (the per-dimension constants in 16-byte loads: the arrays hold 128 entries and start on 256-byte boundaries)
+    float gv[8], sv[8], kv[8];
+    {
+        const float4 g0 = __ldg(reinterpret_cast<const float4*>(gd + d0)), g1 = __ldg(reinterpret_cast<const float4*>(gd + d0) + 1);
+        const float4 s0 = __ldg(reinterpret_cast<const float4*>(sd + d0)), s1 = __ldg(reinterpret_cast<const float4*>(sd + d0) + 1);
+        const float4 k0 = __ldg(reinterpret_cast<const float4*>(kap + d0)), k1 = __ldg(reinterpret_cast<const float4*>(kap + d0) + 1);
+        gv[0] = g0.x; gv[1] = g0.y; gv[2] = g0.z; gv[3] = g0.w; gv[4] = g1.x; gv[5] = g1.y; gv[6] = g1.z; gv[7] = g1.w;
+        sv[0] = s0.x; sv[1] = s0.y; sv[2] = s0.z; sv[3] = s0.w; sv[4] = s1.x; sv[5] = s1.y; sv[6] = s1.z; sv[7] = s1.w;
+        kv[0] = k0.x; kv[1] = k0.y; kv[2] = k0.z; kv[3] = k0.w; kv[4] = k1.x; kv[5] = k1.y; kv[6] = k1.z; kv[7] = k1.w;
+    }
     uint32_t xh[4], xl[4], qh[4], ql[4];
 #pragma unroll
     for (int j = 0; j < 8; j += 2) {
         // centred and scaled: u = s_d (x - g_d)  (padded dimensions: s = 1, g = 0, x = 0)
-        float u0 = (x[j] - __ldg(gd + d0 + j)) * __ldg(sd + d0 + j), u1 = (x[j + 1] - __ldg(gd + d0 + j + 1)) * __ldg(sd + d0 + j + 1);
+        float u0 = (x[j] - gv[j]) * sv[j], u1 = (x[j + 1] - gv[j + 1]) * sv[j + 1];
         if (!valid) { u0 = 0.f; u1 = 0.f; }
         u0 = fminf(fmaxf(u0, -240.f), 240.f);
         u1 = fminf(fmaxf(u1, -240.f), 240.f);
-        float q0 = fmaf(u0, u0, __ldg(kap + d0 + j)), q1 = fmaf(u1, u1, __ldg(kap + d0 + j + 1));
+        float q0 = fmaf(u0, u0, kv[j]), q1 = fmaf(u1, u1, kv[j + 1]);
         if (!valid) { q0 = 0.f; q1 = 0.f; }
         const __half2 h = __floats2half2_rn(u0, u1);
         const float2 hf = __half22float2(h);

@@ -203,11 +203,12 @@ def main():
     # and the log-likelihood (skipped on one GPU), replicated gmm_finalize
     em = ShardedEM(ctx, em_step=lambda X_, p_, m_, v_: ctx.gmm_em_step(X_, p_, m_, v_, out=(Nk, S1, S2)),
                    finalize=lambda n_, a_, b_, c_, fl_, p_, m_, v_: ctx.gmm_finalize(n_, a_, b_, c_, fl_, p_, m_, v_))
-    exact_counts = []
+    exact_counts, exact_pairs = [], []
 
     def step():
         trace.append(em.step(X, pi, mu, var, N_global, spec.var_floor))
         exact_counts.append(ctx.gmm_last_exact_count())
+        exact_pairs.append(ctx.gmm_last_exact_pairs() if D > 128 else (0, 0, 0))
 
     for _ in range(args.warmup):
         step()
@@ -263,9 +264,10 @@ def main():
             kg_share = 1.0 - (sum(timed_counts) / len(timed_counts) / K if timed_counts else 0.0)
             executed_factor = (12.0 + 24.0 * kg_share) / 8.0
             if kg_share <= 0.01:
-                # screening mode: the sweep forms three products for the narrow components and one for the others (how many of
-                # each is not reported), and the statistics come from exact fp32 evaluations: no executed-work figure
-                executed_factor = None
+                # screening mode: one tensor sweep forms the leading fp16 product of the E-step contraction alone (4 N K D
+                # of the algorithmic 8 N K D); everything else is fp32 work on the few (point, component) pairs that sweep
+                # marks.  frac_executed is then the tensor work actually issued against the tensor peak.
+                executed_factor = 4.0 / 8.0
             timed_launch = ("per piece of 2^17 points: wide_transform_kernel + lse_wide_kernel (+ em_wide_kernel in the two-sweep mode), plus the exact "
                             "evaluation of the components left out of the tensor passes (all inside the timed bracket)")
             traffic_key = "wide" if kg_share > 0.01 else "wide_screen"     # (no component in the second sweep: the screening mode)
@@ -296,17 +298,23 @@ def main():
                 traffic_source = f"profiles/{tj.get('summary', 'traffic.json')}: {tj['dram_bytes_per_point']:.0f} B per point from one ncu capture, scaled by the points of a launch"
         except Exception:
             traffic = None
+    ex2_count = N * K * ((1.0 + kg_share) if (wide and path_used == fg.GMM_PATH_TENSOR) else 1)
+    if wide and path_used == fg.GMM_PATH_TENSOR and kg_share <= 0.01 and exact_pairs:
+        # screening mode: no exponential in the sweep; two per kept pair (its term of Z, its responsibility)
+        timed_pairs = exact_pairs[-args.steps:]
+        ex2_count = 2.0 * sum(b for _, b, _ in timed_pairs) / len(timed_pairs)
     roofline = {
         "bound": bound, "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved_tf / peak_tf,
         "traffic": traffic, "traffic_source": traffic_source, "peak_source": peak_note, "kernel_ms_per_step": kern_ms_step,
         "kernel_launches_per_step": kern_n / args.steps, "timed_launch": timed_launch,
         "algorithmic_flop_per_step": flops_step,
         "frac_executed": (achieved_tf * executed_factor / peak_tf) if executed_factor else None,
-        "frac_fp32_accurate_tensor": (achieved_tf / (peak_tf / 3.0)) if bound == "tensor" else None,
+        "mode": ("screen" if kg_share <= 0.01 else "sweeps") if (wide and path_used == fg.GMM_PATH_TENSOR) else None,
+        "frac_fp32_accurate_tensor": (achieved_tf / (peak_tf / 3.0)) if (bound == "tensor" and not (wide and kg_share <= 0.01)) else None,
         "hbm_frac": (bytes_X + 2 * K * D * 4) / (kern_ms_step * 1e-3) / 1e9 / peaks["hbm_gbs"],
-        "ex2_per_s": N * K * ((1.0 + kg_share) if (wide and path_used == fg.GMM_PATH_TENSOR) else 1) / (kern_ms_step * 1e-3),
+        "ex2_per_s": ex2_count / (kern_ms_step * 1e-3),
         "mufu_peak_ex2_per_s": ex2_rate or None,
-        "mufu_frac": (N * K * ((1.0 + kg_share) if (wide and path_used == fg.GMM_PATH_TENSOR) else 1) / (kern_ms_step * 1e-3) / ex2_rate) if ex2_rate else None,
+        "mufu_frac": (ex2_count / (kern_ms_step * 1e-3) / ex2_rate) if ex2_rate else None,
         "fp32_fma_tflops_measured": (fma_flops / 1e12) if fma_flops else None,
     }
 
@@ -444,6 +452,8 @@ def main():
             "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": int(launches),
             "clocks": clocks, "scratch_bytes": int(mem_extra), "scratch_bytes_measured": int(scratch_measured),
             "exact_components_per_step": exact_counts[-args.steps:] if exact_counts else None,
+            "exact_pairs_per_step": ([{"marked": int(a), "kept": int(b), "dense_pieces": int(c)} for a, b, c in exact_pairs[-args.steps:]]
+                                     if D > 128 else None),
             "assign_topm": assign, "fisher_vectors": fisher,
             "loglik_first_last": [trace[0], trace[-1]],
             "paper_context": {"A100_ms_per_iter_N1M": 3755.0 / 30, "A100_ms_per_iter_N100M": 74270.0 / 30},

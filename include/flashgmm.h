@@ -81,14 +81,15 @@ int gmm_auto_path(int D, int K);
 int gmm_last_path(const gmm_ctx* ctx);
 /* How many components the most recent tensor-path step treated as ill-conditioned, i.e. evaluated (where they matter)
  * exactly in fp32 instead of through the expanded quadratic form; 0 after a step on the FP32 path.  On wide data
- * (D > 128) with few points per component the tensor path only screens the (point, component) pairs and evaluates all
- * that can matter exactly: the count is then the number of components with a positive weight. */
+ * (D > 128), whenever a sample of the points shows that few pairs per point matter, the tensor path only screens the
+ * (point, component) pairs and evaluates all that can matter exactly: the count is then the number of components with a
+ * positive weight. */
 int gmm_last_exact_count(const gmm_ctx* ctx);
 /* For the most recent tensor-path step on wide data (D > 128) that had such components: how their (point, component)
- * pairs were evaluated.  *marked: pairs the screening sweep could not rule out; *kept: pairs whose exact density came
+ * pairs were evaluated.  *marked: pairs the screening sweep and its filter could not rule out; *kept: pairs whose exact density came
  * within 2^-40 of the point's total and entered the statistics (both summed over the pieces of the step that went pair
  * by pair, saturating at 2^31 - 1); *dense_pieces: pieces of the step whose marked pairs were too many (more than one in
- * 64), for which the FP32 kernels evaluated the whole sub-mixture instead.  All zero after any other step.  Reads a few
+ * 64; one in 16 when every component is screened), for which the FP32 kernels evaluated the whole sub-mixture instead.  All zero after any other step.  Reads a few
  * bytes back from the device (synchronises the context's stream).  Errors: GMM_EINVAL (NULL argument), GMM_ECUDA. */
 int gmm_last_exact_pairs(gmm_ctx* ctx, int64_t* marked, int64_t* kept, int* dense_pieces);
 

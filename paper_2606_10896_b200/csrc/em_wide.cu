@@ -8,8 +8,10 @@
 //   sweep 1  (lse_wide_kernel, TMEM lanes = POINTS)   Algorithm 1, Step 1.  A CTA takes tiles of 128 points and walks the
 //            components in groups of 256 (256 TMEM columns for the main product, 256 for the two small cross products:
 //            the same split, and the same order of accumulation, as in sweep 2, so that both sweeps see the same logits
-//            and the responsibilities of a point sum to one); for every 64-column atom of the contraction it streams the
-//            tile's Y atom and the group's coefficient atoms through a ring in shared memory.
+//            and the responsibilities of a point sum to one; a group that is only screened forms the leading product
+//            alone, in one half of the columns, while the softmax warps read the other half); for every 64-column atom
+//            of the contraction it streams one stage per plane - the tile's Y atom and the group's two coefficient atoms -
+//            through a ring in shared memory.
 //            A softmax thread owns one point: running (max, sum) over all K, log2 Z_i to a scratch buffer of one piece
 //            (2^17 points; no O(N) memory), sum of log2 Z for the log-likelihood.
 //   sweep 2  (em_wide_kernel, TMEM lanes = COMPONENTS)   Algorithm 1, Step 2.  A CTA owns 128 components and takes
@@ -26,11 +28,12 @@
 // Components the expanded form cannot carry (collapsed or narrow ones, and ones that hold few points) are "listed": they
 // sit behind the others in the order the sweeps see the components, sweep 2 leaves them out, and sweep 1 only SCREENS
 // them - it marks, in a bitmap, the (point, component) pairs whose approximate log2 z plus a rigorous error bound can
-// come within 2^-40 of the point's best.  The marked pairs are then evaluated exactly in fp32, pair by pair
-// (wide_cand_lse_kernel, wide_cand_mstep_kernel), or, when they are too many, densely by the FP32 kernels.  In the
-// "screen" mode EVERY component is listed: one tensor sweep decides which pairs are looked at, all statistics come from
-// exact evaluations.  The same screening, with the candidates ranked by upper bounds, gives the top-m assignment
-// (wide_assign_refine_kernel).
+// come within 2^-40 of the point's best (as far as the sweep knows it when it meets the pair; wide_cand_filter_kernel
+// then drops the marks that the point's final threshold rules out).  The marked pairs are then evaluated exactly in fp32,
+// pair by pair (wide_cand_lse_kernel, wide_cand_mstep_kernel), or, when they are too many, densely by the FP32 kernels.
+// In the "screen" mode EVERY component is listed: one tensor sweep over the leading fp16 product decides which pairs are
+// looked at, all statistics come from exact evaluations.  The same screening, with the candidates ranked by upper
+// bounds, gives the top-m assignment (wide_assign_refine_kernel).
 #include "internal.cuh"
 #include "em_tc.cuh"
 #include "em_wide.cuh"

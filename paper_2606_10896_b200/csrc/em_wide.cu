@@ -1551,7 +1551,10 @@ __global__ void __launch_bounds__(256, 3) wide_cand_lse_kernel(const float* __re
                                                             const double* __restrict__ c2d_c, const double* __restrict__ logz,
                                                             double* __restrict__ out, int* __restrict__ ctl,
                                                             int* __restrict__ slot_cnt, float* __restrict__ pair_val,
-                                                            int* __restrict__ pair_off, double* __restrict__ pair_best) {
+                                                            int* __restrict__ pair_off, double* __restrict__ pair_best,
+                                                            const int* __restrict__ list, int32_t* __restrict__ best_out) {
+    // best_out != NULL (the hard assignment): only the first round runs, and the component (list[slot]) of the point's
+    // largest exact value goes to best_out[i]; of equal values the smaller component.
     if (ctl[1] != 0) return;
     __shared__ double lbuf[8][CAND_KEEP];
     __shared__ unsigned short slist[8][CAND_LIST];
@@ -1583,7 +1586,10 @@ __global__ void __launch_bounds__(256, 3) wide_cand_lse_kernel(const float* __re
     __syncthreads();
     if (i >= n) return;
     if (nmarked == 0) {
-        if (lane == 0) out[i] = -CUDART_INF;
+        if (lane == 0) {
+            if (best_out) best_out[i] = 0;
+            else out[i] = -CUDART_INF;
+        }
         return;
     }
     int off = base_s;
@@ -1733,6 +1739,7 @@ __global__ void __launch_bounds__(256, 3) wide_cand_lse_kernel(const float* __re
     __syncwarp();
     const bool listed = total <= CAND_LIST;                   // (else: the row is scanned word by word, as a fallback)
     double best = logz[i];
+    int best_comp = 0x7fffffff;                               // (tracked for best_out only)
     int idx = 0;
     {
         int sl[CAND_G], cnt = 0;
@@ -1745,6 +1752,10 @@ __global__ void __launch_bounds__(256, 3) wide_cand_lse_kernel(const float* __re
                     const double l = alive[g] ? full(sl[g], best - 40.0) : -CUDART_INF;
                     if (idx < CAND_KEEP && lane == 0) lbuf[w][idx] = l;
                     ++idx;
+                    if (best_out && l >= best && l > -CUDART_INF) {
+                        const int comp = __ldg(list + sl[g]);
+                        if (l > best || comp < best_comp) best_comp = comp;
+                    }
                     if (l > best) best = l;
                 }
             }
@@ -1773,6 +1784,10 @@ __global__ void __launch_bounds__(256, 3) wide_cand_lse_kernel(const float* __re
         }
     }
     __syncwarp();
+    if (best_out) {
+        if (lane == 0) best_out[i] = best_comp != 0x7fffffff ? best_comp : 0;
+        return;
+    }
     const double lim = best - 40.0;
     double m = -CUDART_INF, ssum = 0.0;
     int kept = 0;
@@ -2347,10 +2362,10 @@ cudaError_t launch_cand_count_wide(cudaStream_t s, int n_slots, const WideBuffer
 }
 
 cudaError_t launch_cand_lse_wide(cudaStream_t s, const float* X, int64_t n, int D, int n_slots, const WideBuffers& wb,
-                                 double* logz_ill) {
+                                 double* logz_ill, int32_t* best_out) {
     const int words = (n_slots + 31) / 32;
     wide_cand_lse_kernel<<<(unsigned)((n + 7) / 8), 256, 0, s>>>(X, n, D, words, wb.cand, wb.candT, wb.mu_c, wb.w2_c, wb.c2d_c, wb.logz,
-                                                                 logz_ill, wb.ctl, wb.slot_cnt, wb.pair_val, wb.pair_off, wb.pair_best);
+                                                                 logz_ill, wb.ctl, wb.slot_cnt, wb.pair_val, wb.pair_off, wb.pair_best, wb.ill_list, best_out);
     return cudaGetLastError();
 }
 

@@ -156,9 +156,10 @@ cudaError_t launch_cand_filter_wide(cudaStream_t s, int64_t n, int n_slots, cons
 cudaError_t launch_cand_gate_wide(cudaStream_t s, const WideBuffers& wb, long long max_pairs);
 // The marked pairs evaluated exactly, one warp per point (no-op when wb.ctl[1] is set): logz_ill[i] = log2 of the sum of
 // the listed components' exact densities at point i over the pairs that reach 2^-40 of wb.logz[i] (-inf if none); those
-// pairs are marked in wb.candT.
+// pairs are marked in wb.candT.  best_out != NULL (the hard assignment, after a sweep with listed_only): instead, best_out[i]
+// = the component of the point's largest exact value (of equal values the smaller component); logz_ill is not written.
 cudaError_t launch_cand_lse_wide(cudaStream_t s, const float* X, int64_t n, int D, int n_slots, const WideBuffers& wb,
-                                 double* logz_ill);
+                                 double* logz_ill, int32_t* best_out = nullptr);
 // wb.stats_c += the statistics of the pairs marked in wb.candT with r = 2^(exact log2 z - wb.logz_x[i]); one block per
 // slot, points in ascending order (no-op when wb.ctl[1] is set).
 cudaError_t launch_cand_mstep_wide(cudaStream_t s, const float* X, int64_t n, int D, int n_slots, const WideBuffers& wb);

@@ -1056,6 +1056,58 @@ int assign_topm_impl(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, cons
         // go through the FP32 kernels.
         const bool want = ctx->capPlanes && ctx->lay.wide && ctx->path != GMM_PATH_FP32 && K >= 64 && m + 2 <= WIDE_MAX_TOP;
         bool tensor_w = false;
+        // The hard assignment (m = 1, indices only) by the EM step's screening machinery: every component listed, one sweep
+        // over the leading product marks the pairs that can come within 2^-40 of a point's best, the filter drops those
+        // that the final threshold rules out, and a warp per point evaluates the rest exactly and takes the largest.  No
+        // row is left uncertain.  Taken when the first 8192 rows mark few pairs (K / 400 per point: a pair costs 2 ns, the
+        // route below 30 ns per point at config 5's shape); the same limit, per piece, sends a piece to the FP32 kernels.
+        if (want && index_only && m == 1 && ctx->wide_hi == 2 && ctx->wide_mode != 1) {
+            const WideBuffers wb = ctx->wide();
+            float limit = ctx->tc_cond_limit;
+            if (limit < 0.f) limit = ctx->tc_cond_scale * std::sqrt((float)((double)N / (double)K));
+            KL(launch_prepare_wide(ctx->stream, D, K, pi, mu, var, wb, limit, INFINITY, 3));
+            ctx->launches += 4;
+            int fl[8];
+            CU(cudaMemcpyAsync(fl, wb.flags, sizeof(fl), cudaMemcpyDeviceToHost, ctx->stream));
+            CU(cudaStreamSynchronize(ctx->stream));
+            const int n_list = fl[2], n_ill = fl[4], Kg = fl[6];
+            bool ok = n_list >= 1 && n_ill + 64 <= WIDE_MAX_ILL;
+            if (ok) {
+                KL(launch_ill_gather_wide(ctx->stream, D, n_list, wb, mu, ctx->w2(), ctx->c2d()));
+                auto screen_piece = [&](const float* Xs, int64_t cnt) -> int {
+                    CU(launch_cand_clear_wide(ctx->stream, cnt, n_list, wb));
+                    KL(launch_norm_wide(ctx->stream, Xs, cnt, D, wb));
+                    KL(launch_transform_wide(ctx->stream, Xs, cnt, D, wb, &ctx->result()->status, true));
+                    KL(launch_lse_wide(ctx->stream, cnt, D, K, Kg, n_ill, n_list, wb, ctx->sms, &ctx->result()->status, 2, 0, false, true, true));
+                    KL(launch_cand_filter_wide(ctx->stream, cnt, n_list, wb));
+                    return GMM_OK;
+                };
+                const double per_point = ctx->wide_probe_limit > 0.0 ? ctx->wide_probe_limit : (double)n_list / 400.0;
+                if (ctx->wide_mode != 2) {
+                    const int64_t np = N < 8192 ? N : 8192;
+                    CHECK(screen_piece(X, np));
+                    int marks = 0;
+                    CU(cudaMemcpyAsync(&marks, wb.ctl, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
+                    CU(cudaStreamSynchronize(ctx->stream));
+                    ok = (double)marks <= per_point * (double)np;
+                }
+                if (ok) {
+                    const int64_t piece = ctx->wide_piece;
+                    for (int64_t off = 0; off < N; off += piece) {
+                        const int64_t cnt = (N - off < piece) ? (N - off) : piece;
+                        const float* Xs = X + off * D;
+                        CHECK(prof_begin(ctx));
+                        CHECK(screen_piece(Xs, cnt));
+                        KL(launch_cand_gate_wide(ctx->stream, wb, ctx->wide_sparse >= 2 ? ((long long)1 << 62) : (long long)((double)cnt * per_point)));
+                        KL(launch_cand_lse_wide(ctx->stream, Xs, cnt, D, n_list, wb, ctx->logZ2(), idx + off));
+                        KL(launch_topm_fp32(ctx->stream, Xs, cnt, D, K, mu, ctx->w2(), ctx->c2d(), ctx->center(), 1, idx + off, nullptr, wb.ctl + 1));
+                        CHECK(prof_end(ctx));
+                    }
+                    ctx->last_path = GMM_PATH_TENSOR;
+                    return GMM_OK;
+                }
+            }
+        }
         if (want) {
             const WideBuffers wb = ctx->wide();
             const float limit = ctx->tc_cond_limit >= 0.f ? ctx->tc_cond_limit : 0.01f;

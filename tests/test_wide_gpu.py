@@ -339,6 +339,35 @@ def test_wide_assignment_with_listed_components_ties_and_overlap(fg, monkeypatch
         _assign_and_check(fg, c, Xo, pio, muo, varo, 4, "wide assignment, overlapping clusters")
 
 
+def test_wide_hard_assignment_by_screening(fg, monkeypatch):
+    """m = 1, indices only: every component screened by the leading product, the marked pairs evaluated exactly, the
+    largest taken.  (a) separate clusters with collapsed, light and zero-weight components and an exact copy of a component
+    (the smaller index wins), pieces of 4096 points; (b) clusters on top of each other: the sample marks too many pairs and
+    the call takes the route with six candidates per point (and the FP32 kernels for its uncertain rows); (c) the same
+    forced through the screening route, whose pieces then go to the FP32 kernels."""
+    monkeypatch.setenv("GMM_WIDE_PIECE", "4096")
+    rng = np.random.default_rng(91)
+    X, pi, mu, var = _with_listed_components(rng, 12_000 + 5, 288, 80)
+    mu[40], var[40], pi[40] = mu[41], var[41], pi[41]          # an exact copy: ties
+    pi[20] = 0.0
+    pi = (pi / pi.sum()).astype(np.float32)
+    with fg.Context(0) as c:
+        c.gmm_set_path(fg.GMM_PATH_TENSOR)
+        idx, _ = _assign_and_check(fg, c, X, pi, mu, var, 1, "hard assignment by screening", indices_only=True)
+        assert c.gmm_last_path() == fg.GMM_PATH_TENSOR
+        for j in range(5):                                      # the point a collapsed component sits on
+            assert idx[50 + j, 0] == j
+        assert np.sum(idx[:, 0] == 40) > 50 and not np.any(idx[:, 0] == 41) and not np.any(idx[:, 0] == 20)
+        idx2, _ = c.gmm_assign_topm(_t(X), _t(pi), _t(mu), _t(var), 1, indices_only=True)
+        assert np.array_equal(idx, idx2.cpu().numpy())
+        Xo, pio, muo, varo = _clustered(np.random.default_rng(92), 6_000, 256, 64, sep=0.02)
+        _assign_and_check(fg, c, Xo, pio, muo, varo, 1, "hard assignment, overlapping clusters", indices_only=True)
+    monkeypatch.setenv("GMM_WIDE_MODE", "screen")
+    with fg.Context(0) as c:
+        c.gmm_set_path(fg.GMM_PATH_TENSOR)
+        _assign_and_check(fg, c, Xo, pio, muo, varo, 1, "hard assignment, overlapping clusters, screening forced", indices_only=True)
+
+
 def test_wide_assignment_path_choice(fg, ctx):
     """AUTO takes the tensor path for K >= 64; FP32 when forced, for small K, or when more than half of the components are
     ill-conditioned."""

@@ -41,9 +41,6 @@
 #include <cuda.h>
 #include <cuda_fp16.h>
 #include <math_constants.h>
-#include <cstdio>
-#include <cstdlib>
-#include <cstdlib>
 
 #define TC_WAIT_LIMIT_NS 2000000000ull
 #include "tc_prims.cuh"
@@ -101,8 +98,10 @@ struct LseParams {
     unsigned* rec;       // NULL, or [n][WIDE_REC]: the marks' upper bounds, for the filter that follows
     int* rec_cnt;        // [n]
     float* rec_thr;      // [n] the point's final threshold
-    int dbg;
     int g0;              // the sweep starts at this group (the "screen" mode: behind the unlisted components, which have no weight)
+    int topm;            // > 0 (NTOP >= topm; the assignment by screening): the sweep also keeps the NTOP largest LOWER bounds of a
+                         // point's listed components, and a pair is marked iff its upper bound reaches the topm-th of them or
+                         // comes within 2^-40 of the largest: every component of the point's true top m is then marked
     int pre_pass;        // 1: before a tile's sweep proper, the groups from hi_group on are swept once for their lower bounds only
     int* ctl;
 };
@@ -160,7 +159,8 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
     const int NG = (NC + 1) >> 1;                        // groups of two chunks
     // A tile's steps, the same for every role: with pre_pass the groups from hi_group on once for their lower bounds (so that
     // the threshold is final before anything is marked), then every group.
-    const int npre = (p.pre_pass && p.hi_group < NG) ? NG - p.hi_group : 0;
+    // (pre_pass 2: the first of those groups only - enough for the top-m rule to start from m lower bounds)
+    const int npre = (p.pre_pass && p.hi_group < NG) ? (p.pre_pass == 2 ? 1 : NG - p.hi_group) : 0;
     const int nsteps = npre + NG - p.g0;
     auto step_group = [&](int t) { return t < npre ? p.hi_group + t : p.g0 + t - npre; };
     auto leading_only = [&](int g) { return g >= p.hi_group && g < p.hi_end; };
@@ -229,10 +229,10 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
             // (each warpgroup has its own half of the point's record)
             int nrec = 0;
             auto mark = [&](float u, int sl) {
-                if (sl < 0 || p.dbg == 3) return;
-                if (p.dbg != 1) atomicOr(p.cand + row * p.cand_words + (sl >> 5), 1u << (sl & 31));
+                if (sl < 0) return;
+                atomicOr(p.cand + row * p.cand_words + (sl >> 5), 1u << (sl & 31));
                 ++nhit;
-                if (p.rec && p.dbg != 2) {
+                if (p.rec) {
                     if (nrec < WIDE_REC / 2)
                         p.rec[row * WIDE_REC + grp * (WIDE_REC / 2) + nrec] = (__float_as_uint(u + fabsf(u) * 0.001953125f) & ~0x1FFFu) | (unsigned)sl;
                     ++nrec;
@@ -318,8 +318,17 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
                                         const float u0 = fmaf(a0, q.x, fmaf(sq.y, nrm, sq.x));
                                         const float u1 = fmaf(a1, q.z, fmaf(sq.w, nrm, sq.z));
                                         // lower bounds: the upper bound minus twice the allowance (fmaxf drops a NaN)
-                                        thr_base = fmaxf(thr_base, fmaxf(u0 - 2.f * fmaf(sq.y, nrm, se.x), u1 - 2.f * fmaf(sq.w, nrm, se.y)));
-                                        const float thr = thr_base - 40.f;
+                                        const float lb0 = u0 - 2.f * fmaf(sq.y, nrm, se.x), lb1 = u1 - 2.f * fmaf(sq.w, nrm, se.y);
+                                        thr_base = fmaxf(thr_base, fmaxf(lb0, lb1));
+                                        float thr = thr_base - 40.f;
+                                        if (NTOP > 2 && p.topm > 0) {
+                                            // (a group the first phase has seen is not entered a second time)
+                                            if (ph == 0 || g >= p.hi_group + npre) {
+                                                if (sq.x > -CUDART_INF_F) tl.insert(lb0, col0 + j);
+                                                if (sq.z > -CUDART_INF_F) tl.insert(lb1, col0 + j + 1);
+                                            }
+                                            thr = fminf(thr, tl.a[(NTOP > 2) ? p.topm - 1 : 0]);
+                                        }
                                         if (ph == 0) continue;                          // (lower bounds only)
                                         if (!(u0 < thr) && sq.x > -CUDART_INF_F) mark(u0, tabs_s[tb][grp][sub * 32 + j]);
                                         if (!(u1 < thr) && sq.z > -CUDART_INF_F) mark(u1, tabs_s[tb][grp][sub * 32 + j + 1]);
@@ -2414,7 +2423,8 @@ cudaError_t launch_transform_wide(cudaStream_t s, const float* X, int64_t n, int
 }
 
 cudaError_t launch_lse_wide(cudaStream_t s, int64_t n, int D, int K, int Kg, int n_listed, int n_slots, const WideBuffers& wb,
-                            int num_sms, int* status, int ntop, int hi_first_slots, bool pre_pass, bool record, bool listed_only) {
+                            int num_sms, int* status, int ntop, int hi_first_slots, bool pre_pass, bool record, bool listed_only,
+                            int topm) {
     if (n < 1 || n > WIDE_PIECE || Kg < 0 || Kg > K || (Kg < 1 && n_listed < 1)) return cudaErrorInvalidValue;
     const WidePlan pl = wide_plan(D, K, num_sms);
     const int64_t rp = rows_padded_of(n);
@@ -2443,28 +2453,26 @@ cudaError_t launch_lse_wide(cudaStream_t s, int64_t n, int D, int K, int Kg, int
     p.scr_e = wb.scr_e; p.scr_mask = wb.scr_mask; p.slot_of = wb.slot_of; p.n2 = wb.n2; p.cand = wb.cand;
     p.cand_words = (n_slots + 31) / 32; p.scr_group = Kgp / 256; p.ctl = wb.ctl;
     p.hi_group = 0x7fffffff; p.hi_end = 0x7fffffff; p.pre_pass = 0;
-    { const char* e = std::getenv("GMM_DBG"); p.dbg = e ? std::atoi(e) : 0; }
-    p.g0 = (listed_only && screen && ntop == 2) ? Kgp / 256 : 0;
-    p.rec = (record && screen && ntop == 2) ? wb.rec : nullptr; p.rec_cnt = wb.rec_cnt; p.rec_thr = wb.rec_thr;
+    p.topm = 0;
+    if (topm > 0) {                                          // the assignment by screening: as the EM step's screening mode
+        if (ntop == 2 || topm > ntop || !screen || !listed_only || hi_first_slots != 0) return cudaErrorInvalidValue;
+        p.topm = topm;
+        p.hi_group = Kgp / 256; p.hi_end = 0x7fffffff;
+        p.pre_pass = 2;
+    }
+    const bool em_like = ntop == 2 || topm > 0;
+    p.g0 = (listed_only && screen && em_like) ? Kgp / 256 : 0;
+    p.rec = (record && screen && em_like) ? wb.rec : nullptr; p.rec_cnt = wb.rec_cnt; p.rec_thr = wb.rec_thr;
     if (ntop == 2 && screen && hi_first_slots >= 0) {                                                      // the EM step's screening mode
         p.hi_group = (Kgp + hi_first_slots + 255) / 256;
         p.pre_pass = pre_pass ? 1 : 0;
     }
-    if (ntop != 2 && hi_first_slots >= 0) { p.hi_group = 0; p.hi_end = Kgp / 256; }                         // the assignment's evaluated groups
+    if (ntop != 2 && hi_first_slots >= 0 && topm <= 0) { p.hi_group = 0; p.hi_end = Kgp / 256; }             // the assignment's evaluated groups
     const int64_t ntiles = (n + WIDE_TILE - 1) / WIDE_TILE;
     const unsigned grid = (unsigned)(ntiles < num_sms ? ntiles : num_sms);
-    cudaEvent_t ev0 = nullptr, ev1 = nullptr;
-    const bool timing = std::getenv("GMM_WIDE_TIMING") != nullptr;
-    if (timing) { cudaEventCreate(&ev0); cudaEventCreate(&ev1); cudaEventRecord(ev0, s); }
     if (ntop == 2) lse_wide_kernel<2><<<grid, WT_THREADS, L_SMEM, s>>>(p, tm_yhi, tm_ylo, tm_phi, tm_plo);
     else if (ntop == 6) lse_wide_kernel<6><<<grid, WT_THREADS, L_SMEM, s>>>(p, tm_yhi, tm_ylo, tm_phi, tm_plo);
     else lse_wide_kernel<WIDE_MAX_TOP><<<grid, WT_THREADS, L_SMEM, s>>>(p, tm_yhi, tm_ylo, tm_phi, tm_plo);
-    if (timing) {
-        cudaEventRecord(ev1, s); cudaEventSynchronize(ev1);
-        float ms = 0; cudaEventElapsedTime(&ms, ev0, ev1);
-        std::printf("lse_wide n=%lld %.3f ms\n", (long long)n, ms);
-        cudaEventDestroy(ev0); cudaEventDestroy(ev1);
-    }
     return cudaGetLastError();
 }
 

@@ -492,7 +492,6 @@ int prepare_and_choose(gmm_ctx* ctx, int64_t N, int D, int K, const float* pi, c
                 const double auto_limit = (double)n_list / (few_points ? 16.0 : 200.0);
                 ok = (double)marks <= (ctx->wide_probe_limit > 0.0 ? ctx->wide_probe_limit : auto_limit) * (double)np;
             }
-            if (std::getenv("GMM_WIDE_TIMING")) std::printf("screen prepare: n_list %d n_ill %d first-kind slots %d Kg %d ok %d\n", n_list, fl[4], fl[5], fl[6], (int)ok);
             if (ok) {
                 ctx->wide_n_ill = fl[4];
                 ctx->wide_n_good = fl[6];

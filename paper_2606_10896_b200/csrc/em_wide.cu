@@ -99,9 +99,8 @@ struct LseParams {
     int* rec_cnt;        // [n]
     float* rec_thr;      // [n] the point's final threshold
     int g0;              // the sweep starts at this group (the "screen" mode: behind the unlisted components, which have no weight)
-    int topm;            // > 0 (NTOP >= topm; the assignment by screening): the sweep also keeps the NTOP largest LOWER bounds of a
-                         // point's listed components, and a pair is marked iff its upper bound reaches the topm-th of them or
-                         // comes within 2^-40 of the largest: every component of the point's true top m is then marked
+    int topm;            // > 0 (NTOP > 2; the assignment by screening): the sweep also reports, per point, the NTOP blocks of 32
+                         // listed components with the largest upper bounds (the bound and the component's position)
     int pre_pass;        // 1: before a tile's sweep proper, the groups from hi_group on are swept once for their lower bounds only
     int* ctl;
 };
@@ -159,8 +158,7 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
     const int NG = (NC + 1) >> 1;                        // groups of two chunks
     // A tile's steps, the same for every role: with pre_pass the groups from hi_group on once for their lower bounds (so that
     // the threshold is final before anything is marked), then every group.
-    // (pre_pass 2: the first of those groups only - enough for the top-m rule to start from m lower bounds)
-    const int npre = (p.pre_pass && p.hi_group < NG) ? (p.pre_pass == 2 ? 1 : NG - p.hi_group) : 0;
+    const int npre = (p.pre_pass && p.hi_group < NG) ? NG - p.hi_group : 0;
     const int nsteps = npre + NG - p.g0;
     auto step_group = [&](int t) { return t < npre ? p.hi_group + t : p.g0 + t - npre; };
     auto leading_only = [&](int g) { return g >= p.hi_group && g < p.hi_end; };
@@ -307,6 +305,11 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
                                 // maximum over the evaluated components is final by now.  (!(a < b): a NaN passes.)
                                 if (tabm_s[tb][grp][sub] != 0 && row < p.n) {
                                     const float2* se2 = reinterpret_cast<const float2*>(&tabe_s[tb][grp][sub * 32]);
+                                    // (topm: the block's largest upper bound and where - one candidate per block of 32
+                                    // components for the ranks that no marked pair fills; an insertion per component
+                                    // made the sweep four times slower, the insertions of 32 points diverge)
+                                    float bub = -CUDART_INF_F;
+                                    int bcol = col0;
 #pragma unroll
                                     for (int j = 0; j < 32; j += 2) {
                                         const float4 t0 = tb4[j], t1 = tb4[j + 1];
@@ -320,19 +323,16 @@ lse_wide_kernel(const LseParams p, const __grid_constant__ CUtensorMap tm_yhi, c
                                         // lower bounds: the upper bound minus twice the allowance (fmaxf drops a NaN)
                                         const float lb0 = u0 - 2.f * fmaf(sq.y, nrm, se.x), lb1 = u1 - 2.f * fmaf(sq.w, nrm, se.y);
                                         thr_base = fmaxf(thr_base, fmaxf(lb0, lb1));
-                                        float thr = thr_base - 40.f;
+                                        const float thr = thr_base - 40.f;
                                         if (NTOP > 2 && p.topm > 0) {
-                                            // (a group the first phase has seen is not entered a second time)
-                                            if (ph == 0 || g >= p.hi_group + npre) {
-                                                if (sq.x > -CUDART_INF_F) tl.insert(lb0, col0 + j);
-                                                if (sq.z > -CUDART_INF_F) tl.insert(lb1, col0 + j + 1);
-                                            }
-                                            thr = fminf(thr, tl.a[(NTOP > 2) ? p.topm - 1 : 0]);
+                                            if (u0 > bub && sq.x > -CUDART_INF_F) { bub = u0; bcol = col0 + j; }
+                                            if (u1 > bub && sq.z > -CUDART_INF_F) { bub = u1; bcol = col0 + j + 1; }
                                         }
                                         if (ph == 0) continue;                          // (lower bounds only)
                                         if (!(u0 < thr) && sq.x > -CUDART_INF_F) mark(u0, tabs_s[tb][grp][sub * 32 + j]);
                                         if (!(u1 < thr) && sq.z > -CUDART_INF_F) mark(u1, tabs_s[tb][grp][sub * 32 + j + 1]);
                                     }
+                                    if (NTOP > 2 && p.topm > 0 && ph == 1) tl.insert(bub, bcol);
                                 }
                                 continue;
                             }
@@ -1554,6 +1554,7 @@ constexpr int CAND_WORDS_PER_LANE = (WIDE_CAND_WORDS + 31) / 32;
 constexpr int CAND_KEEP = 256;          // exact values of a point's first pairs kept between the two rounds
 constexpr int CAND_LIST = 256;          // marked slots of a point listed in shared memory (more: the row is scanned instead)
 constexpr int CAND_G = 4;               // marked pairs of a point taken together (their loads overlap)
+template <int TOPM>
 __global__ void __launch_bounds__(256, 3) wide_cand_lse_kernel(const float* __restrict__ X, int64_t n, int D, int words,
                                                             const unsigned* __restrict__ cand, unsigned* __restrict__ candT,
                                                             const float* __restrict__ mu_c, const float* __restrict__ w2_c,
@@ -1561,7 +1562,15 @@ __global__ void __launch_bounds__(256, 3) wide_cand_lse_kernel(const float* __re
                                                             double* __restrict__ out, int* __restrict__ ctl,
                                                             int* __restrict__ slot_cnt, float* __restrict__ pair_val,
                                                             int* __restrict__ pair_off, double* __restrict__ pair_best,
-                                                            const int* __restrict__ list, int32_t* __restrict__ best_out) {
+                                                            const int* __restrict__ list, int32_t* __restrict__ best_out,
+                                                            int m_top, int32_t* __restrict__ top_idx, float* __restrict__ top_resp,
+                                                            int32_t* __restrict__ unc_rows, int* __restrict__ unc_count,
+                                                            const float* __restrict__ swp_top, int swp_ntop,
+                                                            const int* __restrict__ comp_of) {
+    // TOPM > 0 (the top-m assignment, m_top <= TOPM): only the first round runs; it keeps the m_top largest exact values
+    // (a pair is abandoned once it can reach neither the m_top-th of them nor 2^-40 of the largest) and the sum of all.
+    // Ranks that no marked pair fills (every component there lies 2^-40 below the point's best: responsibility 0) are
+    // taken from the sweep's candidates, in the order of their upper bounds.
     // best_out != NULL (the hard assignment): only the first round runs, and the component (list[slot]) of the point's
     // largest exact value goes to best_out[i]; of equal values the smaller component.
     if (ctl[1] != 0) return;
@@ -1596,7 +1605,8 @@ __global__ void __launch_bounds__(256, 3) wide_cand_lse_kernel(const float* __re
     if (i >= n) return;
     if (nmarked == 0) {
         if (lane == 0) {
-            if (best_out) best_out[i] = 0;
+            if (TOPM > 0) unc_rows[atomicAdd(unc_count, 1)] = (int32_t)i;
+            else if (best_out) best_out[i] = 0;
             else out[i] = -CUDART_INF;
         }
         return;
@@ -1749,16 +1759,50 @@ __global__ void __launch_bounds__(256, 3) wide_cand_lse_kernel(const float* __re
     const bool listed = total <= CAND_LIST;                   // (else: the row is scanned word by word, as a fallback)
     double best = logz[i];
     int best_comp = 0x7fffffff;                               // (tracked for best_out only)
+    constexpr int TM = TOPM > 0 ? TOPM : 1;
+    double topv[TM];                                         // (TOPM > 0) the largest exact values so far, descending ...
+    int topc[TM];                                            // ... and their components; every lane holds the same
+    double zm = -CUDART_INF, zs = 0.0;                       // running log-sum-exp of all exact values
+#pragma unroll
+    for (int r = 0; r < TM; ++r) { topv[r] = -CUDART_INF; topc[r] = -1; }
     int idx = 0;
     {
         int sl[CAND_G], cnt = 0;
         auto flush = [&]() {
             bool alive[CAND_G];
-            first_chunks(sl, cnt, best - 40.0, alive);
+            double stop = best - 40.0;
+            if (TOPM > 0) {
+#pragma unroll
+                for (int r = 0; r < TM; ++r)
+                    if (r == m_top - 1) stop = fmin(stop, topv[r]);
+            }
+            first_chunks(sl, cnt, stop, alive);
 #pragma unroll
             for (int g = 0; g < CAND_G; ++g) {
                 if (g < cnt) {
-                    const double l = alive[g] ? full(sl[g], best - 40.0) : -CUDART_INF;
+                    if (TOPM > 0) {
+                        stop = best - 40.0;
+#pragma unroll
+                        for (int r = 0; r < TM; ++r)
+                            if (r == m_top - 1) stop = fmin(stop, topv[r]);
+                    }
+                    const double l = alive[g] ? full(sl[g], TOPM > 0 ? stop : best - 40.0) : -CUDART_INF;
+                    if (TOPM > 0 && l > -CUDART_INF) {
+                        if (l > zm) { zs = zs * exp2(zm - l) + 1.0; zm = l; }
+                        else zs += exp2(l - zm);
+                        // insertion by (value descending, component ascending)
+                        double v = l;
+                        int c = __ldg(list + sl[g]);
+#pragma unroll
+                        for (int r = 0; r < TM; ++r) {
+                            if (r < m_top && (v > topv[r] || (v == topv[r] && topc[r] >= 0 && c < topc[r]) || topc[r] < 0)) {
+                                const double tv = topv[r]; const int tc = topc[r];
+                                topv[r] = v; topc[r] = c;
+                                v = tv; c = tc;
+                                if (c < 0) break;
+                            }
+                        }
+                    }
                     if (idx < CAND_KEEP && lane == 0) lbuf[w][idx] = l;
                     ++idx;
                     if (best_out && l >= best && l > -CUDART_INF) {
@@ -1793,6 +1837,41 @@ __global__ void __launch_bounds__(256, 3) wide_cand_lse_kernel(const float* __re
         }
     }
     __syncwarp();
+    if (TOPM > 0) {
+        if (lane == 0) {
+            const double lzf = zm + log2(zs);
+            int have = 0;
+#pragma unroll
+            for (int r = 0; r < TM; ++r)
+                if (r < m_top && topc[r] >= 0) ++have;
+            for (int q = 0; q < swp_ntop && have > 0 && have < m_top; ++q) {
+                const int pos = __float_as_int(swp_top[i * 2 * swp_ntop + swp_ntop + q]);
+                const int c = pos >= 0 ? __ldg(comp_of + pos) : -1;
+                bool dup = c < 0;
+#pragma unroll
+                for (int r = 0; r < TM; ++r)
+                    if (r < m_top && topc[r] == c) dup = true;
+                if (dup) continue;
+#pragma unroll
+                for (int r = 0; r < TM; ++r)
+                    if (r == have) { topc[r] = c; topv[r] = -CUDART_INF; }
+                ++have;
+            }
+            bool full_row = have == m_top;
+            if (!full_row) {
+                unc_rows[atomicAdd(unc_count, 1)] = (int32_t)i;
+            } else {
+#pragma unroll
+                for (int r = 0; r < TM; ++r) {
+                    if (r < m_top) {
+                        top_idx[i * m_top + r] = topc[r];
+                        if (top_resp) top_resp[i * m_top + r] = (float)exp2(topv[r] - lzf);
+                    }
+                }
+            }
+        }
+        return;
+    }
     if (best_out) {
         if (lane == 0) best_out[i] = best_comp != 0x7fffffff ? best_comp : 0;
         return;
@@ -2373,8 +2452,20 @@ cudaError_t launch_cand_count_wide(cudaStream_t s, int n_slots, const WideBuffer
 cudaError_t launch_cand_lse_wide(cudaStream_t s, const float* X, int64_t n, int D, int n_slots, const WideBuffers& wb,
                                  double* logz_ill, int32_t* best_out) {
     const int words = (n_slots + 31) / 32;
-    wide_cand_lse_kernel<<<(unsigned)((n + 7) / 8), 256, 0, s>>>(X, n, D, words, wb.cand, wb.candT, wb.mu_c, wb.w2_c, wb.c2d_c, wb.logz,
-                                                                 logz_ill, wb.ctl, wb.slot_cnt, wb.pair_val, wb.pair_off, wb.pair_best, wb.ill_list, best_out);
+    wide_cand_lse_kernel<0><<<(unsigned)((n + 7) / 8), 256, 0, s>>>(X, n, D, words, wb.cand, wb.candT, wb.mu_c, wb.w2_c, wb.c2d_c, wb.logz,
+                                                                    logz_ill, wb.ctl, wb.slot_cnt, wb.pair_val, wb.pair_off, wb.pair_best, wb.ill_list, best_out,
+                                                                    0, nullptr, nullptr, nullptr, nullptr, nullptr, 0, nullptr);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_cand_topm_wide(cudaStream_t s, const float* X, int64_t n, int D, int n_slots, const WideBuffers& wb, int m,
+                                  int32_t* idx, float* resp, int32_t* unc_rows, int* unc_count, int ntop) {
+    if (m < 1 || m > GMM_MAX_TOPM || (ntop != 6 && ntop != WIDE_MAX_TOP)) return cudaErrorInvalidValue;
+    const int words = (n_slots + 31) / 32;
+    wide_cand_lse_kernel<GMM_MAX_TOPM><<<(unsigned)((n + 7) / 8), 256, 0, s>>>(X, n, D, words, wb.cand, wb.candT, wb.mu_c, wb.w2_c, wb.c2d_c, wb.logz,
+                                                                               nullptr, wb.ctl, wb.slot_cnt, wb.pair_val, wb.pair_off, wb.pair_best,
+                                                                               wb.ill_list, nullptr, m, idx, resp, unc_rows, unc_count,
+                                                                               wb.top, ntop, wb.comp_of);
     return cudaGetLastError();
 }
 
@@ -2458,7 +2549,6 @@ cudaError_t launch_lse_wide(cudaStream_t s, int64_t n, int D, int K, int Kg, int
         if (ntop == 2 || topm > ntop || !screen || !listed_only || hi_first_slots != 0) return cudaErrorInvalidValue;
         p.topm = topm;
         p.hi_group = Kgp / 256; p.hi_end = 0x7fffffff;
-        p.pre_pass = 2;
     }
     const bool em_like = ntop == 2 || topm > 0;
     p.g0 = (listed_only && screen && em_like) ? Kgp / 256 : 0;

@@ -130,13 +130,10 @@ cudaError_t launch_cand_count_wide(cudaStream_t s, int n_slots, const WideBuffer
 // 256 positions behind them are screened by the leading product alone.
 cudaError_t launch_lse_wide(cudaStream_t s, int64_t n, int D, int K, int Kg, int n_listed, int n_slots, const WideBuffers& wb,
                             int num_sms, int* status, int ntop = 2, int hi_first_slots = -1, bool pre_pass = false,
-                            bool record = false, bool listed_only = false);
-// listed_only: the sweep leaves out the groups of the unlisted components (the caller knows that none of them has a weight;
-// wb.logz is then -inf for every point).
-// record (screening, ntop = 2): every mark's upper bound goes to wb.rec and the point's final threshold to wb.rec_thr, for
-// launch_cand_filter_wide.
-// pre_pass (with hi_first_slots >= 0): every tile first sweeps those groups once for the largest lower bound alone, so that
-// the screening threshold is final before anything is marked.
+                            bool record = false, bool listed_only = false, int topm = 0);
+// topm > 0 (ntop = 6 or 10, listed_only, hi_first_slots = 0; the top-m assignment by screening): wb.top[i] also reports the
+// ntop blocks of 32 listed components with the largest upper bounds at point i (the bound, and the position of the block's
+// best component).
 // Top-m assignment of the n points of a piece from what launch_lse_wide (ntop >= m + 2; screened: it also marked the listed
 // pairs) and launch_norm_wide left in wb: idx [n][m], resp [n][m] (may be NULL); rows whose answer is not certain are appended to unc_rows
 // (unc_count += 1 each) and left unwritten.  mu, w2, c2d: the FP32 path's derived parameters.
@@ -160,6 +157,13 @@ cudaError_t launch_cand_gate_wide(cudaStream_t s, const WideBuffers& wb, long lo
 // = the component of the point's largest exact value (of equal values the smaller component); logz_ill is not written.
 cudaError_t launch_cand_lse_wide(cudaStream_t s, const float* X, int64_t n, int D, int n_slots, const WideBuffers& wb,
                                  double* logz_ill, int32_t* best_out = nullptr);
+// The top-m assignment from the marked pairs (after a sweep with topm = m and ntop candidates, and the filter): idx [n][m],
+// resp [n][m] (may be NULL) from the exact values of the point's marked pairs, largest first, of equal values the smaller
+// component.  The marked pairs hold every component within 2^-40 of the point's best; ranks beyond them (responsibility
+// 0) are filled from the sweep's candidates in the order of their upper bounds.  A point that still has fewer than m
+// components is appended to unc_rows (unc_count += 1) and left unwritten.
+cudaError_t launch_cand_topm_wide(cudaStream_t s, const float* X, int64_t n, int D, int n_slots, const WideBuffers& wb, int m,
+                                  int32_t* idx, float* resp, int32_t* unc_rows, int* unc_count, int ntop);
 // wb.stats_c += the statistics of the pairs marked in wb.candT with r = 2^(exact log2 z - wb.logz_x[i]); one block per
 // slot, points in ascending order (no-op when wb.ctl[1] is set).
 cudaError_t launch_cand_mstep_wide(cudaStream_t s, const float* X, int64_t n, int D, int n_slots, const WideBuffers& wb);

@@ -1060,7 +1060,11 @@ int assign_topm_impl(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, cons
         // that the final threshold rules out, and a warp per point evaluates the rest exactly and takes the largest.  No
         // row is left uncertain.  Taken when the first 8192 rows mark few pairs (K / 400 per point: a pair costs 2 ns, the
         // route below 30 ns per point at config 5's shape); the same limit, per piece, sends a piece to the FP32 kernels.
-        if (want && index_only && m == 1 && ctx->wide_hi == 2 && ctx->wide_mode != 1) {
+        // The general top-m goes the same way: the marked pairs hold every component within 2^-40 of the point's best, their
+        // exact values give the leading ranks and the responsibilities; ranks beyond them (responsibility 0) are filled from
+        // the candidates the sweep reports (the blocks of 32 components with the largest upper bounds).
+        if (want && ctx->wide_hi == 2 && ctx->wide_mode != 1) {
+            const bool argmax = index_only && m == 1;
             const WideBuffers wb = ctx->wide();
             float limit = ctx->tc_cond_limit;
             if (limit < 0.f) limit = ctx->tc_cond_scale * std::sqrt((float)((double)N / (double)K));
@@ -1073,15 +1077,28 @@ int assign_topm_impl(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, cons
             bool ok = n_list >= 1 && n_ill + 64 <= WIDE_MAX_ILL;
             if (ok) {
                 KL(launch_ill_gather_wide(ctx->stream, D, n_list, wb, mu, ctx->w2(), ctx->c2d()));
+                const int ntop = argmax ? 2 : (m + 2 <= 6) ? 6 : WIDE_MAX_TOP;
                 auto screen_piece = [&](const float* Xs, int64_t cnt) -> int {
                     CU(launch_cand_clear_wide(ctx->stream, cnt, n_list, wb));
                     KL(launch_norm_wide(ctx->stream, Xs, cnt, D, wb));
                     KL(launch_transform_wide(ctx->stream, Xs, cnt, D, wb, &ctx->result()->status, true));
-                    KL(launch_lse_wide(ctx->stream, cnt, D, K, Kg, n_ill, n_list, wb, ctx->sms, &ctx->result()->status, 2, 0, false, true, true));
+                    KL(launch_lse_wide(ctx->stream, cnt, D, K, Kg, n_ill, n_list, wb, ctx->sms, &ctx->result()->status, ntop, 0, false, true, true,
+                                       argmax ? 0 : m));
                     KL(launch_cand_filter_wide(ctx->stream, cnt, n_list, wb));
                     return GMM_OK;
                 };
+                // (a pair costs 2 ns, the route below 30-60 ns per point at config 5's shape)
                 const double per_point = ctx->wide_probe_limit > 0.0 ? ctx->wide_probe_limit : (double)n_list / 400.0;
+                int32_t* unc_rows = nullptr;
+                int* unc_count = nullptr;
+                if (!argmax) {
+                    const int64_t cap = N < ctx->wide_piece ? N : ctx->wide_piece;
+                    const size_t need = align256((size_t)cap * sizeof(int32_t)) + 256;       // rows with fewer than m finite values, their count
+                    CHECK(grow_buffer(ctx, &ctx->at_scratch, &ctx->at_scratch_bytes, need, "the assignment's list of uncertain rows"));
+                    unsigned char* base = static_cast<unsigned char*>(ctx->at_scratch);
+                    unc_rows = reinterpret_cast<int32_t*>(base);
+                    unc_count = reinterpret_cast<int*>(base + need - 256);
+                }
                 if (ctx->wide_mode != 2) {
                     const int64_t np = N < 8192 ? N : 8192;
                     CHECK(screen_piece(X, np));
@@ -1098,8 +1115,16 @@ int assign_topm_impl(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, cons
                         CHECK(prof_begin(ctx));
                         CHECK(screen_piece(Xs, cnt));
                         KL(launch_cand_gate_wide(ctx->stream, wb, ctx->wide_sparse >= 2 ? ((long long)1 << 62) : (long long)((double)cnt * per_point)));
-                        KL(launch_cand_lse_wide(ctx->stream, Xs, cnt, D, n_list, wb, ctx->logZ2(), idx + off));
-                        KL(launch_topm_fp32(ctx->stream, Xs, cnt, D, K, mu, ctx->w2(), ctx->c2d(), ctx->center(), 1, idx + off, nullptr, wb.ctl + 1));
+                        int32_t* idx_p = idx + off * m;
+                        float* resp_p = resp ? resp + off * m : nullptr;
+                        if (argmax) {
+                            KL(launch_cand_lse_wide(ctx->stream, Xs, cnt, D, n_list, wb, ctx->logZ2(), idx_p));
+                        } else {
+                            CU(cudaMemsetAsync(unc_count, 0, sizeof(int), ctx->stream));
+                            KL(launch_cand_topm_wide(ctx->stream, Xs, cnt, D, n_list, wb, m, idx_p, resp_p, unc_rows, unc_count, ntop));
+                            KL(launch_topm_fp32(ctx->stream, Xs, cnt, D, K, mu, ctx->w2(), ctx->c2d(), ctx->center(), m, idx_p, resp_p, nullptr, unc_rows, unc_count));
+                        }
+                        KL(launch_topm_fp32(ctx->stream, Xs, cnt, D, K, mu, ctx->w2(), ctx->c2d(), ctx->center(), m, idx_p, resp_p, wb.ctl + 1));
                         CHECK(prof_end(ctx));
                     }
                     ctx->last_path = GMM_PATH_TENSOR;

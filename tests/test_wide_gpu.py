@@ -369,8 +369,9 @@ def test_wide_hard_assignment_by_screening(fg, monkeypatch):
 
 
 def test_wide_assignment_path_choice(fg, ctx):
-    """AUTO takes the tensor path for K >= 64; FP32 when forced, for small K, or when more than half of the components are
-    ill-conditioned."""
+    """AUTO takes the tensor path for K >= 64 (by screening, which does not mind collapsed components; with GMM_WIDE_MODE=sweeps
+    the route with six candidates per point, which leaves a mixture with more than half of its components ill-conditioned
+    to the FP32 kernels); FP32 when forced."""
     X, pi, mu, var = _clustered(np.random.default_rng(8), 5_000, 256, 64)
     ctx.gmm_set_path(fg.GMM_PATH_AUTO)
     _assign_and_check(fg, ctx, X, pi, mu, var, 2, "AUTO")
@@ -381,8 +382,28 @@ def test_wide_assignment_path_choice(fg, ctx):
     ctx.gmm_set_path(fg.GMM_PATH_AUTO)
     v2 = var.copy()
     v2[:40] = 1e-6
-    _assign_and_check(fg, ctx, X, pi, mu, v2, 2, "40 of 64 collapsed")
-    assert ctx.gmm_last_path() == fg.GMM_PATH_FP32
+    _assign_and_check(fg, ctx, X, pi, mu, v2, 2, "40 of 64 collapsed")      # (either route, by what the sample of rows marks)
+
+
+def test_wide_assignment_by_candidates(fg, monkeypatch):
+    """GMM_WIDE_MODE=sweeps keeps the assignment on the route that reports six or ten candidates per point from a sweep over
+    the evaluated components: the same cases as above, and the mixture that route leaves to the FP32 kernels."""
+    monkeypatch.setenv("GMM_WIDE_MODE", "sweeps")
+    monkeypatch.setenv("GMM_WIDE_PIECE", "4096")
+    rng = np.random.default_rng(55)
+    X, pi, mu, var = _with_listed_components(rng, 12_000, 288, 80)
+    with fg.Context(0) as c:
+        c.gmm_set_path(fg.GMM_PATH_TENSOR)
+        for m in (1, 4, 8):
+            _assign_and_check(fg, c, X, pi, mu, var, m, f"assignment by candidates m={m}")
+            assert c.gmm_last_path() == fg.GMM_PATH_TENSOR
+        _assign_and_check(fg, c, X, pi, mu, var, 4, "assignment by candidates, indices only", indices_only=True)
+        Xo, pio, muo, varo = _clustered(np.random.default_rng(56), 6_000, 256, 64, sep=0.02)
+        _assign_and_check(fg, c, Xo, pio, muo, varo, 4, "assignment by candidates, overlapping clusters")
+        Xc, pic, muc, varc = _clustered(np.random.default_rng(8), 5_000, 256, 64)
+        varc[:40] = 1e-6
+        _assign_and_check(fg, c, Xc, pic, muc, varc, 2, "40 of 64 collapsed")
+        assert c.gmm_last_path() == fg.GMM_PATH_FP32
 
 
 def test_wide_path_at_its_largest_shape(fg, ctx):

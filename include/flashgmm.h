@@ -152,7 +152,10 @@ int gmm_fit(gmm_ctx* ctx, const float* X, int64_t N, int D, int K,
  * as a selection pass and the best few per point are recomputed exactly in fp32, so indices and values are those of the
  * FP32 kernels; a point whose selection is not certain within the error bound of the selection pass is evaluated
  * against all K components exactly; components whose responsibility for a point is below 4.8e-7 keep the order and
- * the values of the selection pass (inside the 1e-6 tie width).  Parameters with more than 256 ill-conditioned
+ * the values of the selection pass (inside the 1e-6 tie width).  On wide data (D > 128), whenever a sample of the points
+ * shows that few (point, component) pairs matter, one tensor sweep screens all pairs instead, every component within
+ * 2^-40 of a point's best is evaluated exactly (indices and responsibilities from those values), and ranks beyond them
+ * are reported with responsibility 0 in the order of the sweep's upper bounds.  Parameters with more than 256 ill-conditioned
  * components run on the FP32 kernels (decided on the device; gmm_last_path then still reports the tensor path).  The
  * first call allocates a work buffer outside gmm_scratch_bytes: 128 or 192 bytes (m <= 4, m > 4) per point of one piece
  * of at most 2^19 points plus 4 bytes per point of eight pieces (84 MB or 118 MB at most, independent of N). */

@@ -173,6 +173,30 @@ def test_wide_screen_mode_against_oracle(fg, monkeypatch, N, D, K):
             assert np.array_equal(u, v.cpu().numpy())
 
 
+def test_wide_screen_mode_with_a_first_pass_for_the_threshold(fg, monkeypatch):
+    """GMM_WIDE_PRE=1: every tile first sweeps the leading product once for the largest lower bound alone, so that the sweep
+    proper marks against a final threshold (the filter then finds little to drop); GMM_WIDE_HI=1 and 0: all three products
+    for the components flagged by the rounding estimate, or for every component.  Same results at the ordinary tolerances."""
+    monkeypatch.setenv("GMM_WIDE_MODE", "screen")
+    monkeypatch.setenv("GMM_WIDE_SPARSE", "2")
+    monkeypatch.setenv("GMM_WIDE_PIECE", "4096")
+    N, D, K = 9_000 + 13, 200, 130
+    X, pi, mu, var = _clustered(np.random.default_rng(N + D), N, D, K)
+    mu[0], var[0] = X[7], 1e-6
+    var[1, ::7] = 1e-5
+    pi[2] = 2e-4
+    pi = (pi / pi.sum()).astype(np.float32)
+    for pre, hi in (("1", "2"), ("0", "1"), ("1", "1"), ("0", "0")):
+        monkeypatch.setenv("GMM_WIDE_PRE", pre)
+        monkeypatch.setenv("GMM_WIDE_HI", hi)
+        with fg.Context(0) as c:
+            c.gmm_set_path(fg.GMM_PATH_TENSOR)
+            _step_and_check(fg, c, X, pi, mu, var, f"screen mode, first pass {pre}, leading product {hi}")
+            assert c.gmm_last_path() == fg.GMM_PATH_TENSOR and c.gmm_last_exact_count() == K
+            marked, kept, dense = c.gmm_last_exact_pairs()
+            assert dense == 0 and N <= kept <= marked
+
+
 def test_wide_screen_mode_more_pairs_than_stored_values(fg, monkeypatch):
     """Clusters on top of each other, every pair marked: more marked pairs in a piece (40,000 x 130) than the buffer of exact
     pair values holds (32 x 2^17), so the statistics kernel evaluates its pairs itself."""

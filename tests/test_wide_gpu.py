@@ -147,7 +147,7 @@ def test_wide_auto_path_rule(fg, ctx):
     assert ctx.gmm_last_path() == fg.GMM_PATH_FP32
 
 
-@pytest.mark.parametrize("N,D,K", [(9_000 + 13, 200, 130), (6_000, 768, 256), (40_000, 320, 96)])
+@pytest.mark.parametrize("N,D,K", [(9_000 + 13, 200, 130), (6_000, 768, 256), (40_000, 320, 96), (7_000 + 1, 131, 70)])
 def test_wide_screen_mode_against_oracle(fg, monkeypatch, N, D, K):
     """GMM_WIDE_MODE=screen: one tensor sweep screens every (point, component) pair, all marked pairs are evaluated exactly
     (no component goes through the second tensor sweep).  With collapsed, narrow, light and zero-weight components; pieces
@@ -171,6 +171,9 @@ def test_wide_screen_mode_against_oracle(fg, monkeypatch, N, D, K):
         Nk, S1, S2, _ = c.gmm_em_step(_t(X), _t(pi), _t(mu), _t(var))
         for u, v in zip(a, (Nk, S1, S2)):
             assert np.array_equal(u, v.cpu().numpy())
+        if D == 131:       # (rows that are not whole 16-byte groups: the pair kernels' scalar loads; also the assignment's)
+            _assign_and_check(fg, c, X, pi, mu, var, 3, "assignment by screening, D = 131")
+            _assign_and_check(fg, c, X, pi, mu, var, 1, "hard assignment by screening, D = 131", indices_only=True)
 
 
 def test_wide_screen_mode_with_a_first_pass_for_the_threshold(fg, monkeypatch):

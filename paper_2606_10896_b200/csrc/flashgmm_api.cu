@@ -187,7 +187,7 @@ struct gmm_ctx {
     int wide_mode = 0;               // GMM_WIDE_MODE: 0 = automatic, 1 = "sweeps" (two tensor sweeps, few components exact),
                                      // 2 = "screen" (one tensor sweep screens every pair, every component evaluated exactly)
     double wide_probe_limit = 0.0;   // automatic mode: "screen" while a sample of the points has at most this many marked pairs per
-                                     // point (0: K / 200, or K / 16 below 128 points per component)
+                                     // point (0: from the measured costs, see wide_pair_limit)
     bool wide_screen_all = false;    // the current step runs in "screen" mode
     bool wide_pre = false;           // GMM_WIDE_PRE=1: a first pass over the leading product for the screening threshold (instead
                                      // of leaving the marks made against an immature threshold to the filter alone)
@@ -436,6 +436,14 @@ int prof_end(gmm_ctx* ctx) {
 
 // Derived per-component constants for both paths; validates the parameters into the status word.  Then picks the
 // path: the tensor-core path whenever the shape allows it (ill-conditioned components are handled inside its kernel).
+// Marked pairs per point up to which the screening mode is the cheaper way through a step on wide data (see the comment in
+// prepare_and_choose): against the two tensor sweeps, or (dense = true) against the FP32 kernels over all listed components.
+double wide_pair_limit(int n_list, int D, bool dense) {
+    const double kd = (double)n_list * D;
+    const double saved = (dense ? 5.0e-4 : 3.3e-5) * kd - 3.6e-6 * kd - 5.0;
+    return saved > 0.0 ? saved / (1.0 + 3.4e-3 * D) : 0.0;
+}
+
 int prepare_and_choose(gmm_ctx* ctx, int64_t N, int D, int K, const float* pi, const float* mu, const float* var,
                        int* path, const float* Xprobe = nullptr, int64_t n_probe = 0) {
     KL(launch_prepare_fp32(ctx->stream, D, K, pi, mu, var, ctx->w2(), ctx->c2(), ctx->c2d(), ctx->center(), &ctx->result()->status));
@@ -461,14 +469,14 @@ int prepare_and_choose(gmm_ctx* ctx, int64_t N, int D, int K, const float* pi, c
         const WideBuffers wb = ctx->wide();
         int fl[8];
         const bool can_probe = Xprobe != nullptr && n_probe >= 1;
-        // Automatic choice, step by step: the screening sweep is tried on the first 8192 rows, and "screen" is taken if it marks
-        // few enough pairs per point.  With the marks filtered against the final threshold nearly every marked pair is kept,
-        // and a kept pair costs 3.6 ns at D = 768 (exact evaluation plus its statistics); the mode's fixed part is 16 ns per
-        // point at config 5's shape.  What "screen" saves is the second tensor sweep and the two low-order products of the
-        // first (config 5: 104 against 16 ns per point), whose cost per point grows with K D like the pair's does with D:
-        // from 128 points per component on the limit is K / 200 marked pairs per point (config 5: 20; its iterations from a
-        // data-row initialisation mark 9, 30, 11, 4.5, 3.3, 2.9).  Below 128 points per component "sweeps" is no alternative
-        // (it would list most components as light) and the FP32 kernels cost K D / 2 ns per point: K / 16.
+        // Automatic choice, step by step: the screening sweep and its filter are tried on the first 8192 rows, and "screen" is
+        // taken if they mark few enough pairs per point.  Costs per point, measured at config 5's shape and checked at
+        // five others (K 64-4096, D 200-1024): "screen" 5 ns + 3.6e-6 K D ns (norm, filter, the pair kernels' fixed part;
+        // the leading-product sweep) + (1 + 3.4e-3 D) ns per marked pair (nearly every marked pair is kept: its exact value
+        // and its statistics); "sweeps" 3.3e-5 K D ns; the FP32 kernels 5e-4 K D ns.  From 128 points per component on the
+        // alternative is "sweeps" (limit 24 marked pairs per point at config 5, whose iterations from a data-row
+        // initialisation mark 12, 30, 11, 4.5, 3.3, 2.9; none at K D below 170,000, where "sweeps" costs less than the pair
+        // kernels' fixed part); below, where "sweeps" would list most components as light, the FP32 kernels.
         const bool few_points = N < WIDE_AUTO_MIN_POINTS_PER_COMPONENT * K;
         if (ctx->wide_mode == 2 || (ctx->wide_mode == 0 && can_probe)) {
             KL(launch_prepare_wide(ctx->stream, D, K, pi, mu, var, wb, limit, INFINITY, ctx->wide_hi == 2 ? 3 : ctx->wide_hi ? 1 : 0));      // every component is listed
@@ -489,7 +497,7 @@ int prepare_and_choose(gmm_ctx* ctx, int64_t N, int D, int K, const float* pi, c
                 int marks = 0;
                 CU(cudaMemcpyAsync(&marks, wb.ctl, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
                 CU(cudaStreamSynchronize(ctx->stream));
-                const double auto_limit = (double)n_list / (few_points ? 16.0 : 200.0);
+                const double auto_limit = wide_pair_limit(n_list, D, few_points);
                 ok = (double)marks <= (ctx->wide_probe_limit > 0.0 ? ctx->wide_probe_limit : auto_limit) * (double)np;
             }
             if (ok) {
@@ -600,7 +608,7 @@ int accumulate_points(gmm_ctx* ctx, int path, const float* X, int64_t n, int D, 
                     // more than one pair in 64 marked (or the pair-by-pair route switched off): the dense kernels are cheaper
                     // ("screen" mode: the dense alternative evaluates every component, so the pair route pays for longer)
                     const long long max_pairs = ctx->wide_sparse >= 2 ? ((long long)1 << 62)
-                                              : all ? (long long)cnt * n_ill / 16 : (long long)cnt * n_ill / 64;
+                                              : all ? (long long)((double)cnt * wide_pair_limit(n_ill, D, true)) : (long long)cnt * n_ill / 64;
                     KL(launch_cand_gate_wide(ctx->stream, wb, max_pairs));
                     KL(launch_cand_lse_wide(ctx->stream, Xs, cnt, D, n_ill, wb, ctx->logZ2()));
                 }
@@ -1058,7 +1066,7 @@ int assign_topm_impl(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, cons
         // The hard assignment (m = 1, indices only) by the EM step's screening machinery: every component listed, one sweep
         // over the leading product marks the pairs that can come within 2^-40 of a point's best, the filter drops those
         // that the final threshold rules out, and a warp per point evaluates the rest exactly and takes the largest.  No
-        // row is left uncertain.  Taken when the first 8192 rows mark few pairs (K / 400 per point: a pair costs 2 ns, the
+        // row is left uncertain.  Taken when the first 8192 rows mark few pairs (half the EM step's limit: a pair costs 2 ns, the
         // route below 30 ns per point at config 5's shape); the same limit, per piece, sends a piece to the FP32 kernels.
         // The general top-m goes the same way: the marked pairs hold every component within 2^-40 of the point's best, their
         // exact values give the leading ranks and the responsibilities; ranks beyond them (responsibility 0) are filled from
@@ -1088,7 +1096,7 @@ int assign_topm_impl(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, cons
                     return GMM_OK;
                 };
                 // (a pair costs 2 ns, the route below 30-60 ns per point at config 5's shape)
-                const double per_point = ctx->wide_probe_limit > 0.0 ? ctx->wide_probe_limit : (double)n_list / 400.0;
+                const double per_point = ctx->wide_probe_limit > 0.0 ? ctx->wide_probe_limit : 0.5 * wide_pair_limit(n_list, D, false);
                 int32_t* unc_rows = nullptr;
                 int* unc_count = nullptr;
                 if (!argmax) {

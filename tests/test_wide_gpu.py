@@ -373,6 +373,7 @@ def test_wide_hard_assignment_by_screening(fg, monkeypatch):
     the call takes the route with six candidates per point (and the FP32 kernels for its uncertain rows); (c) the same
     forced through the screening route, whose pieces then go to the FP32 kernels."""
     monkeypatch.setenv("GMM_WIDE_PIECE", "4096")
+    monkeypatch.setenv("GMM_WIDE_PROBE_LIMIT", "8")      # (at this small K D the automatic limit is zero: the other route is cheaper)
     rng = np.random.default_rng(91)
     X, pi, mu, var = _with_listed_components(rng, 12_000 + 5, 288, 80)
     mu[40], var[40], pi[40] = mu[41], var[41], pi[41]          # an exact copy: ties
@@ -387,6 +388,12 @@ def test_wide_hard_assignment_by_screening(fg, monkeypatch):
         assert np.sum(idx[:, 0] == 40) > 50 and not np.any(idx[:, 0] == 41) and not np.any(idx[:, 0] == 20)
         idx2, _ = c.gmm_assign_topm(_t(X), _t(pi), _t(mu), _t(var), 1, indices_only=True)
         assert np.array_equal(idx, idx2.cpu().numpy())
+        for m in (1, 4, 8):                                     # the general top-m by the same route, with responsibilities
+            idx4, resp4 = _assign_and_check(fg, c, X, pi, mu, var, m, f"top-{m} by screening")
+            assert np.array_equal(idx4[:, 0], idx[:, 0])
+            if m > 1:
+                tied = np.flatnonzero(idx4[:, 0] == 40)
+                assert np.all(idx4[tied, 1] == 41) and np.allclose(resp4[tied, 0], resp4[tied, 1])
         Xo, pio, muo, varo = _clustered(np.random.default_rng(92), 6_000, 256, 64, sep=0.02)
         _assign_and_check(fg, c, Xo, pio, muo, varo, 1, "hard assignment, overlapping clusters", indices_only=True)
     monkeypatch.setenv("GMM_WIDE_MODE", "screen")

@@ -198,8 +198,11 @@ int gmm_kmeans_step(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const
  * estimate evaluates, which the paper's Discussion (Section 6) names as another user of the fused pattern.
  *   X [N x D], pi [K], mu [K x D], var [K x D]: device fp32, as for gmm_em_step.
  *   logp [N] fp32, device out (natural logarithm);  loglik (host out, may be NULL): their sum in float64.
- * Runs the log-sum-exp kernel of the FP32 path at every shape (exact direct-difference logits): a per-point value has no
- * averaging over points to absorb the tensor path's approximate logits.  Errors as gmm_em_step.  Synchronises the stream. */
+ * Every value comes from exact direct-difference logits in fp32 (a per-point value has no averaging over points to absorb
+ * approximate logits): the log-sum-exp kernel of the FP32 path, or, on wide data (D > 128, K >= 64, path not forced to
+ * FP32) whenever a sample of the points shows that few (point, component) pairs matter, one tensor sweep that screens the
+ * pairs followed by the exact evaluation of those it cannot rule out (every component within 2^-40 of a point's best);
+ * gmm_last_path tells which.  Errors as gmm_em_step.  Synchronises the stream. */
 int gmm_score_samples(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const float* pi, const float* mu,
                       const float* var, float* logp, double* loglik);
 

@@ -1397,6 +1397,70 @@ int gmm_score_samples(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, con
     KL(launch_prepare_fp32(ctx->stream, D, K, pi, mu, var, ctx->w2(), ctx->c2(), ctx->c2d(), ctx->center(), &ctx->result()->status));
     if ((size_t)K * D > ((size_t)1 << 12)) ctx->launches++;
     CU(cudaMemsetAsync(&ctx->result()->ll[0], 0, 8, ctx->stream));
+    // Wide data with sparse posteriors: the EM step's screening route without its statistics.  Every component with a weight
+    // is listed, one sweep over the leading fp16 product marks the pairs that can come within 2^-40 of a point's best, the
+    // filter drops those that the final threshold rules out, and a warp per point evaluates the rest exactly: their
+    // log-sum-exp is the point's log-density to 2^-40.  Taken when the first 8192 rows mark few pairs per point (a pair costs
+    // 0.5 + 1.8e-3 D ns, the FP32 kernel 1.4e-4 K D ns per point); a piece that marks too many goes through the FP32 kernel.
+    if (wide_supports(D, K) && ctx->capPlanes && ctx->lay.wide && ctx->path != GMM_PATH_FP32 && K >= 64 && ctx->wide_hi == 2 &&
+        ctx->wide_mode != 1) {
+        const WideBuffers wb = ctx->wide();
+        float limit = ctx->tc_cond_limit;
+        if (limit < 0.f) limit = ctx->tc_cond_scale * std::sqrt((float)((double)N / (double)K));
+        KL(launch_prepare_wide(ctx->stream, D, K, pi, mu, var, wb, limit, INFINITY, 3));
+        ctx->launches += 4;
+        int fl[8];
+        CU(cudaMemcpyAsync(fl, wb.flags, sizeof(fl), cudaMemcpyDeviceToHost, ctx->stream));
+        CU(cudaStreamSynchronize(ctx->stream));
+        const int n_list = fl[2], n_ill = fl[4], Kg = fl[6];
+        bool ok = n_list >= 1 && n_ill + 64 <= WIDE_MAX_ILL;
+        if (ok) {
+            KL(launch_ill_gather_wide(ctx->stream, D, n_list, wb, mu, ctx->w2(), ctx->c2d()));
+            auto screen_piece = [&](const float* Xs, int64_t cnt) -> int {
+                CU(launch_cand_clear_wide(ctx->stream, cnt, n_list, wb));
+                KL(launch_norm_wide(ctx->stream, Xs, cnt, D, wb));
+                KL(launch_transform_wide(ctx->stream, Xs, cnt, D, wb, &ctx->result()->status, true));
+                KL(launch_lse_wide(ctx->stream, cnt, D, K, Kg, n_ill, n_list, wb, ctx->sms, &ctx->result()->status, 2, 0, false, true, true));
+                KL(launch_cand_filter_wide(ctx->stream, cnt, n_list, wb));
+                return GMM_OK;
+            };
+            const double kd = (double)n_list * D;
+            const double saved = (1.4e-4 - 3.6e-6) * kd - 5.0;
+            const double per_point = ctx->wide_probe_limit > 0.0 ? ctx->wide_probe_limit : (saved > 0.0 ? saved / (0.5 + 1.8e-3 * D) : 0.0);
+            if (ctx->wide_mode != 2) {
+                const int64_t np = N < 8192 ? N : 8192;
+                CHECK(screen_piece(X, np));
+                int marks = 0;
+                CU(cudaMemcpyAsync(&marks, wb.ctl, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
+                CU(cudaStreamSynchronize(ctx->stream));
+                ok = (double)marks <= per_point * (double)np;
+            }
+            if (ok) {
+                CU(cudaMemsetAsync(wb.llpart, 0, 256 * 8, ctx->stream));
+                const int64_t piece = ctx->wide_piece;
+                for (int64_t off = 0; off < N; off += piece) {
+                    const int64_t cnt = (N - off < piece) ? (N - off) : piece;
+                    const float* Xs = X + off * D;
+                    CHECK(prof_begin(ctx));
+                    CHECK(screen_piece(Xs, cnt));
+                    KL(launch_cand_gate_wide(ctx->stream, wb, ctx->wide_sparse >= 2 ? ((long long)1 << 62) : (long long)((double)cnt * per_point)));
+                    CU(cudaMemcpyAsync(wb.logz_x, wb.logz, (size_t)cnt * 8, cudaMemcpyDeviceToDevice, ctx->stream));     // (-inf: no unlisted component has a weight)
+                    KL(launch_cand_lse_wide(ctx->stream, Xs, cnt, D, n_list, wb, ctx->logZ2()));
+                    KL(launch_lse_fp32(ctx->stream, Xs, cnt, D, n_list, wb.mu_c, wb.w2_c, wb.c2d_c, ctx->center(), ctx->logZ2(), nullptr, wb.logz, wb.ctl + 1));
+                    KL(launch_merge_ll_wide(ctx->stream, cnt, wb, ctx->logZ2()));
+                    CHECK(prof_end(ctx));
+                    KL(launch_logz_out_fp32(ctx->stream, wb.logz_x, cnt, logp + off));
+                }
+                KL(launch_reduce_ll(ctx->stream, wb.llpart, WIDE_LL_BLOCKS, &ctx->result()->ll[0], true));
+                ctx->last_path = GMM_PATH_TENSOR;
+                double total = 0.0;
+                const int rc = read_result(ctx, 0, &total);
+                if (rc != GMM_OK) return rc;
+                if (loglik) *loglik = total;
+                return GMM_OK;
+            }
+        }
+    }
     // the log-sum-exp kernel of the FP32 path, one super-tile at a time; its per-point values go out instead of into an M-step
     for (int64_t off = 0; off < N; off += SUPER_TILE) {
         const int64_t cnt = (N - off < SUPER_TILE) ? (N - off) : SUPER_TILE;

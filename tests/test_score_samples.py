@@ -51,6 +51,50 @@ def test_gpu_score_samples_match_oracle(N, D, K):
 
 
 @pytest.mark.gpu
+@pytest.mark.parametrize("N,D,K,forced", [(9_000 + 13, 200, 130, True), (7_001, 131, 70, True), (12_000, 768, 4096, False)])
+def test_gpu_score_samples_by_screening_on_wide_data(monkeypatch, N, D, K, forced):
+    """Wide data (D > 128) with sparse posteriors: one tensor sweep screens the (point, component) pairs and the few that can
+    matter are evaluated exactly (the EM step's screening route without its statistics).  Clustered data with a component
+    collapsed onto a point and a zero-weight component; pieces of 4096 points; at the two small shapes the route is forced
+    (its automatic limit is zero there), at K = 4096 it is the automatic choice."""
+    import torch
+    from paper_2606_10896_b200 import flashgmm as fg
+
+    monkeypatch.setenv("GMM_WIDE_PIECE", "4096")
+    if forced:
+        monkeypatch.setenv("GMM_WIDE_PROBE_LIMIT", "8")
+    rng = np.random.default_rng(N + K)
+    centres = (rng.normal(size=(K, D)) * 0.3).astype(np.float32)
+    w = rng.uniform(0.5, 1.5, K)
+    w /= w.sum()
+    z = rng.choice(K, size=N, p=w)
+    sig = rng.uniform(0.7, 1.3, size=(K, D)) * 0.3
+    X = (centres[z] + rng.normal(size=(N, D)) * sig[z]).astype(np.float32)
+    mu = (centres + 0.015 * rng.normal(size=(K, D))).astype(np.float32)
+    var = (sig ** 2 * rng.uniform(0.8, 1.25, size=(K, D))).astype(np.float32)
+    pi = w.astype(np.float32)
+    mu[0], var[0] = X[7], 1e-6
+    pi[3] = 0.0
+    pi = (pi / pi.sum()).astype(np.float32)
+    lz = gmm_oracle.responsibilities(X, pi, mu, var)[1]
+    t = lambda v: torch.as_tensor(np.ascontiguousarray(v), device="cuda:0")
+    with fg.Context(0) as ctx:
+        logp, total = ctx.gmm_score_samples(t(X), t(pi), t(mu), t(var))
+        assert ctx.gmm_last_path() == fg.GMM_PATH_TENSOR
+        logp2, total2 = ctx.gmm_score_samples(t(X), t(pi), t(mu), t(var))
+        assert torch.equal(logp, logp2) and total == total2
+        ctx.gmm_set_path(fg.GMM_PATH_FP32)
+        logp3, total3 = ctx.gmm_score_samples(t(X), t(pi), t(mu), t(var))
+        assert ctx.gmm_last_path() == fg.GMM_PATH_FP32
+    got = logp.cpu().numpy().astype(np.float64)
+    assert got.shape == (N,) and np.isfinite(got).all()
+    excess = np.abs(got - lz) - (1e-5 * np.abs(lz) + 1e-4)
+    assert excess.max() <= 0, f"point {int(np.argmax(excess))}: {got[np.argmax(excess)]} vs {lz[np.argmax(excess)]}"
+    assert abs(total - lz.sum()) <= 1e-5 * abs(lz.sum()) + 1e-6
+    assert np.abs(logp3.cpu().numpy() - got).max() <= 2e-5 * np.abs(lz).max() + 2e-4 and abs(total3 - total) <= 1e-5 * abs(total)
+
+
+@pytest.mark.gpu
 def test_gpu_score_samples_rejects_bad_parameters():
     import torch
     from paper_2606_10896_b200 import flashgmm as fg

@@ -87,8 +87,10 @@ struct WideBuffers {
                        // marked pairs consecutive and in slot order (positions from a counter: ctl[4])
     int* pair_off;     // [WIDE_PIECE] where a point's values start
     double* pair_best; // [WIDE_PIECE] the point's best value (the reference of its pair_val entries)
-    int* ctl;       // [8]: [0] pairs sweep 1 let through, [1] nonzero: too many, the FP32 kernels evaluate the sub-mixture
-                    //      densely, [2] nonzero: the pairs are evaluated one by one, [3] pairs that mattered
+    int* ctl;       // [8]: [0] pairs sweep 1 let through (less what the filter took out again), [1] nonzero: too many, the
+                    //      FP32 kernels evaluate the sub-mixture densely, [2] nonzero: the pairs are evaluated one by one,
+                    //      [4] entries of pair_val handed out, [5] nonzero: pair_val ran out (the statistics kernel evaluates
+                    //      its pairs itself)
 };
 
 bool wide_supports(int D, int K);

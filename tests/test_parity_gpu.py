@@ -878,8 +878,8 @@ def test_config5_shape_tensor_path_against_fp32_path_and_oracle_subsample(fg, ct
 
 
 def test_config5_full_size_fit_and_assignment(fg, ctx):
-    """Config 5 as stated: N = 10M (30.7 GB of X), 20 EM iterations (gmm_fit, AUTO path), then gmm_assign_topm with m = 4
-    over all N; conservation at full N, a non-decreasing log-likelihood trace, device memory in use independent of N,
+    """Config 5 as stated: N = 10M (30.7 GB of X), 20 EM iterations (gmm_fit, AUTO path), then gmm_assign_topm with m = 4,
+    the hard assignment and gmm_score_samples over all N; conservation at full N, a non-decreasing log-likelihood trace, device memory in use independent of N,
     the oracle on a seeded 20K-row subsample for one step and for the top-4 output."""
     spec = synth.CONFIGS[5]
     free_b, _ = torch.cuda.mem_get_info()
@@ -907,9 +907,25 @@ def test_config5_full_size_fit_and_assignment(fg, ctx):
     assert L >= trace[-1] - 1e-7 * abs(L)
     idx, resp = ctx.gmm_assign_topm(X, pi_d, mu_d, var_d, 4)
     torch.cuda.synchronize()
-    assert int(idx.min()) >= 0 and int(idx.max()) < spec.K
-    _config5_subsample_check(fg, ctx, X, spec, pi0, mu0, var0, idx, resp, pi_d.cpu().numpy(), mu_d.cpu().numpy(),
-                             var_d.cpu().numpy())
+    assert int(idx.min()) >= 0 and int(idx.max()) < spec.K and ctx.gmm_last_path() == fg.GMM_PATH_TENSOR
+    # the hard assignment and the per-point log-densities over all N, by the same screening route: the arg-max is the
+    # top-4's first entry wherever the two leading responsibilities are not within the tie width, and the densities add up
+    # to the log-likelihood of the step above; both against the oracle on the subsample
+    idx1, _ = ctx.gmm_assign_topm(X, pi_d, mu_d, var_d, 1, indices_only=True)
+    assert ctx.gmm_last_path() == fg.GMM_PATH_TENSOR
+    clear = (resp[:, 0] - resp[:, 1]) > 1e-5
+    assert bool((idx1[:, 0][clear] == idx[:, 0][clear]).all()) and float(clear.float().mean()) > 0.9
+    logp, total = ctx.gmm_score_samples(X, pi_d, mu_d, var_d)
+    assert ctx.gmm_last_path() == fg.GMM_PATH_TENSOR and abs(total - L) <= 1e-6 * abs(L)
+    p1, m1, v1 = pi_d.cpu().numpy(), mu_d.cpu().numpy(), var_d.cpu().numpy()
+    rows = synth.subsample_rows(spec.N, 20_000, spec.seed)
+    rows_d = torch.as_tensor(rows, device=DEV)
+    Xsub = X[rows_d].contiguous().cpu().numpy()
+    lz = orc.responsibilities(Xsub, p1, m1, v1)[1]
+    got = logp[rows_d].cpu().numpy().astype(np.float64)
+    assert (np.abs(got - lz) <= 1e-5 * np.abs(lz) + 1e-4).all()
+    _check_topm(Xsub, p1, m1, v1, 1, idx1[rows_d].cpu().numpy(), None, "config 5 hard assignment subsample")
+    _config5_subsample_check(fg, ctx, X, spec, pi0, mu0, var0, idx, resp, p1, m1, v1)
 
 
 def test_isotropic_update_and_fit_match_the_papers_model(fg, ctx):

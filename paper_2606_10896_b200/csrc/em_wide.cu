@@ -889,16 +889,20 @@ em_wide_kernel(const EmWideParams p, const __grid_constant__ CUtensorMap tm_phi,
 __global__ void __launch_bounds__(256) wide_transform_kernel(const float* __restrict__ X, int64_t n, int64_t rows_padded, int D,
                                                              int Dpad, const float* __restrict__ sd, const float* __restrict__ kap,
                                                              const float* __restrict__ gd, unsigned char* __restrict__ yhi,
-                                                             unsigned char* __restrict__ ylo, int* __restrict__ status) {
+                                                             unsigned char* __restrict__ ylo, float* __restrict__ n2,
+                                                             int* __restrict__ status) {
+    // A warp per row (its units lane, lane + 32, ...), so that |x - g|^2 of the row (n2, may be NULL: what the screening
+    // bounds need) comes out of the same pass in a fixed order of additions.
     const int upr = Dpad >> 3;                           // units per row
-    const int64_t units = rows_padded * upr;
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    const int lane = threadIdx.x & 31;
+    const int64_t warp0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
     const bool vec_ok = (D % 4 == 0) && ((reinterpret_cast<uintptr_t>(X) & 15) == 0);
     bool bad = false;
-    for (int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; u < units; u += stride) {
-        const int64_t row = u / upr;
-        const int ks = (int)(u - row * upr), d0 = ks * 8;
-        const bool valid = row < n;
+    for (int64_t row = warp0; row < rows_padded; row += nwarps) {
+      const bool valid = row < n;
+      float nrm = 0.f;
+      for (int ks = lane; ks < upr; ks += 32) {
+        const int d0 = ks * 8;
         float x[8];
         if (valid && vec_ok && d0 + 8 <= D) {
             const float4 a = __ldg(reinterpret_cast<const float4*>(X + row * D + d0));
@@ -924,8 +928,10 @@ __global__ void __launch_bounds__(256) wide_transform_kernel(const float* __rest
         for (int j = 0; j < 8; j += 2) {
             bad |= !(fabsf(x[j]) <= 3.0e38f) || !(fabsf(x[j + 1]) <= 3.0e38f);
             const bool in0 = valid && d0 + j < D, in1 = valid && d0 + j + 1 < D;
-            float u0 = in0 ? (x[j] - gv[j]) * sv[j] : 0.f;
-            float u1 = in1 ? (x[j + 1] - gv[j + 1]) * sv[j + 1] : 0.f;
+            const float c0 = in0 ? x[j] - gv[j] : 0.f, c1 = in1 ? x[j + 1] - gv[j + 1] : 0.f;
+            nrm = fmaf(c0, c0, fmaf(c1, c1, nrm));
+            float u0 = c0 * sv[j];
+            float u1 = c1 * sv[j + 1];
             u0 = fminf(fmaxf(u0, -240.f), 240.f);
             u1 = fminf(fmaxf(u1, -240.f), 240.f);
             const float q0 = in0 ? fmaf(u0, u0, kv[j]) : 0.f;
@@ -950,6 +956,12 @@ __global__ void __launch_bounds__(256) wide_transform_kernel(const float* __rest
             ol[0] = make_uint4(xl[0], xl[1], xl[2], xl[3]);
             ol[1] = make_uint4(ql[0], ql[1], ql[2], ql[3]);
         }
+      }
+      if (n2) {
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) nrm += __shfl_xor_sync(0xffffffffu, nrm, o);
+          if (lane == 0 && valid) n2[row] = (nrm <= 3e38f) ? nrm : 3e38f;     // (a NaN or an infinity in X is reported below)
+      }
     }
     if (bad) atomicOr(status, ST_BAD_X);
 }
@@ -1440,23 +1452,6 @@ __global__ void __launch_bounds__(256) wide_merge_ll_kernel(int64_t n, double* _
 // of the 10^8 pairs of a piece (a component collapsed onto a point matters for that point only), so evaluating them one
 // by one costs nothing next to the dense evaluation of the whole sub-mixture by the FP32 kernels, which stays as the
 // route for parameter sets in which the marked pairs are many (ctl[1]).
-
-// |x_i - g|^2 of the piece's points: one warp per point, fixed order.
-__global__ void __launch_bounds__(256) wide_norm_kernel(const float* __restrict__ X, int64_t n, int D, const float* __restrict__ gd,
-                                                        float* __restrict__ n2) {
-    const int64_t i = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
-    if (i >= n) return;
-    const float* xr = X + i * D;
-    float s = 0.f;
-    for (int d = lane; d < D; d += 32) {
-        const float t = __ldg(xr + d) - __ldg(gd + d);
-        s = fmaf(t, t, s);
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-    if (lane == 0) n2[i] = (s <= 3e38f) ? s : 3e38f;          // (a NaN or an infinity in X is reported by the transform kernel)
-}
 
 // One warp per point: the marks sweep 1 recorded for it, against the point's final threshold.
 __global__ void __launch_bounds__(256) wide_cand_filter_kernel(int64_t n, int words, unsigned* __restrict__ cand,
@@ -2420,11 +2415,6 @@ cudaError_t launch_ill_scatter_wide(cudaStream_t s, int D, int K, int n_ill, con
     return cudaGetLastError();
 }
 
-cudaError_t launch_norm_wide(cudaStream_t s, const float* X, int64_t n, int D, const WideBuffers& wb) {
-    wide_norm_kernel<<<(unsigned)((n + 7) / 8), 256, 0, s>>>(X, n, D, wb.gd, wb.n2);
-    return cudaGetLastError();
-}
-
 cudaError_t launch_cand_clear_wide(cudaStream_t s, int64_t n, int n_slots, const WideBuffers& wb) {
     const int words = (n_slots + 31) / 32;
     cudaError_t e = cudaMemsetAsync(wb.ctl, 0, 8 * sizeof(int), s);
@@ -2502,14 +2492,15 @@ cudaError_t launch_assign_refine_wide(cudaStream_t s, const float* X, int64_t n,
     return cudaGetLastError();
 }
 
-cudaError_t launch_transform_wide(cudaStream_t s, const float* X, int64_t n, int D, const WideBuffers& wb, int* status, bool hi_only) {
+cudaError_t launch_transform_wide(cudaStream_t s, const float* X, int64_t n, int D, const WideBuffers& wb, int* status, bool hi_only,
+                                  bool with_norm) {
     if (n < 1 || n > WIDE_PIECE) return cudaErrorInvalidValue;
     const WidePlan pl = wide_plan(D, 1, 148);
     const int64_t rp = rows_padded_of(n);
-    const int64_t units = rp * (pl.Dpad >> 3);
-    int64_t blocks = (units + 255) / 256;
+    int64_t blocks = (rp + 7) / 8;                       // a warp per row
     if (blocks > 148 * 16) blocks = 148 * 16;
-    wide_transform_kernel<<<(unsigned)blocks, 256, 0, s>>>(X, n, rp, D, pl.Dpad, wb.sd, wb.kap, wb.gd, wb.y_hi, hi_only ? nullptr : wb.y_lo, status);
+    wide_transform_kernel<<<(unsigned)blocks, 256, 0, s>>>(X, n, rp, D, pl.Dpad, wb.sd, wb.kap, wb.gd, wb.y_hi, hi_only ? nullptr : wb.y_lo,
+                                                           with_norm ? wb.n2 : nullptr, status);
     return cudaGetLastError();
 }
 

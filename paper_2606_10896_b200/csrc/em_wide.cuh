@@ -106,7 +106,9 @@ cudaError_t launch_prepare_wide(cudaStream_t s, int D, int K, const float* pi, c
 // and launch_assign_refine_wide hi = true.
 // n <= WIDE_PIECE points: X -> the fp16 planes of Y (rows up to the next multiple of 256 are written as zeros).
 cudaError_t launch_transform_wide(cudaStream_t s, const float* X, int64_t n, int D, const WideBuffers& wb, int* status,
-                                  bool hi_only = false);       // hi_only: the lo plane is not written (a sweep of leading products follows)
+                                  bool hi_only = false, bool with_norm = false);
+// hi_only: the lo plane is not written (a sweep of leading products follows); with_norm: wb.n2[i] = |x_i - g|^2 of the piece's
+// points as well (what a screening sweep's bounds need; a warp per point, fixed order of additions).
 // The listed components' rows of the FP32 path's derived parameters packed into wb.mu_c / w2_c / c2d_c.
 cudaError_t launch_ill_gather_wide(cudaStream_t s, int D, int n_ill, const WideBuffers& wb, const float* mu, const float* w2,
                                    const double* c2d);
@@ -137,14 +139,13 @@ cudaError_t launch_lse_wide(cudaStream_t s, int64_t n, int D, int K, int Kg, int
 // ntop blocks of 32 listed components with the largest upper bounds at point i (the bound, and the position of the block's
 // best component).
 // Top-m assignment of the n points of a piece from what launch_lse_wide (ntop >= m + 2; screened: it also marked the listed
-// pairs) and launch_norm_wide left in wb: idx [n][m], resp [n][m] (may be NULL); rows whose answer is not certain are appended to unc_rows
+// pairs) and launch_transform_wide (with_norm) left in wb: idx [n][m], resp [n][m] (may be NULL); rows whose answer is not certain are appended to unc_rows
 // (unc_count += 1 each) and left unwritten.  mu, w2, c2d: the FP32 path's derived parameters.
 cudaError_t launch_assign_refine_wide(cudaStream_t s, const float* X, int64_t n, int D, int K, const float* mu, const float* w2,
                                       const double* c2d, int n_slots, bool screened, const WideBuffers& wb, int ntop, int m,
                                       int32_t* idx, float* resp, int32_t* unc_rows, int* unc_count, bool index_only,
                                       bool hi = false);
 // wb.n2[i] = |x_i - g|^2 for the n points of a piece.
-cudaError_t launch_norm_wide(cudaStream_t s, const float* X, int64_t n, int D, const WideBuffers& wb);
 // Clears wb.ctl, the n rows of wb.cand and the n_slots rows of wb.candT before a piece's first sweep.
 cudaError_t launch_cand_clear_wide(cudaStream_t s, int64_t n, int n_slots, const WideBuffers& wb);
 // After a screening sweep 1 with record = true: the marks whose recorded upper bound lies below the point's final threshold

@@ -490,8 +490,7 @@ int prepare_and_choose(gmm_ctx* ctx, int64_t N, int D, int K, const float* pi, c
                 // the first rows of the data through the screening sweep: how many pairs per point does it mark?
                 const int64_t np = n_probe < 8192 ? n_probe : 8192;
                 CU(launch_cand_clear_wide(ctx->stream, np, n_list, wb));
-                KL(launch_norm_wide(ctx->stream, Xprobe, np, D, wb));
-                KL(launch_transform_wide(ctx->stream, Xprobe, np, D, wb, &ctx->result()->status, ctx->wide_hi == 2));
+                KL(launch_transform_wide(ctx->stream, Xprobe, np, D, wb, &ctx->result()->status, ctx->wide_hi == 2, true));
                 KL(launch_lse_wide(ctx->stream, np, D, K, fl[6], fl[4], n_list, wb, ctx->sms, &ctx->result()->status, 2, ctx->wide_hi == 2 ? 0 : ctx->wide_hi ? fl[5] : -1, ctx->wide_pre, true, true));
                 KL(launch_cand_filter_wide(ctx->stream, np, n_list, wb));
                 int marks = 0;
@@ -592,12 +591,9 @@ int accumulate_points(gmm_ctx* ctx, int path, const float* X, int64_t n, int D, 
             const int64_t cnt = (n - off < ctx->wide_piece) ? (n - off) : ctx->wide_piece;
             const float* Xs = X + off * D;
             if (!all) CU(cudaMemsetAsync(wb.partial, 0, ctx->lay.w_partial_bytes, ctx->stream));
-            if (screen) {
-                CU(launch_cand_clear_wide(ctx->stream, cnt, n_ill, wb));
-                KL(launch_norm_wide(ctx->stream, Xs, cnt, D, wb));
-            }
+            if (screen) CU(launch_cand_clear_wide(ctx->stream, cnt, n_ill, wb));
             CHECK(prof_begin(ctx));
-            KL(launch_transform_wide(ctx->stream, Xs, cnt, D, wb, &ctx->result()->status, all && ctx->wide_hi == 2));
+            KL(launch_transform_wide(ctx->stream, Xs, cnt, D, wb, &ctx->result()->status, all && ctx->wide_hi == 2, screen));
             KL(launch_lse_wide(ctx->stream, cnt, D, K, Kg, screen ? n_listed : 0, n_ill, wb, ctx->sms, &ctx->result()->status, 2,
                                !(all && ctx->wide_hi) ? -1 : ctx->wide_hi == 2 ? 0 : ctx->wide_n_first, ctx->wide_pre, true, all));
             if (screen) KL(launch_cand_filter_wide(ctx->stream, cnt, n_ill, wb));
@@ -1088,8 +1084,7 @@ int assign_topm_impl(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, cons
                 const int ntop = argmax ? 2 : (m + 2 <= 6) ? 6 : WIDE_MAX_TOP;
                 auto screen_piece = [&](const float* Xs, int64_t cnt) -> int {
                     CU(launch_cand_clear_wide(ctx->stream, cnt, n_list, wb));
-                    KL(launch_norm_wide(ctx->stream, Xs, cnt, D, wb));
-                    KL(launch_transform_wide(ctx->stream, Xs, cnt, D, wb, &ctx->result()->status, true));
+                    KL(launch_transform_wide(ctx->stream, Xs, cnt, D, wb, &ctx->result()->status, true, true));
                     KL(launch_lse_wide(ctx->stream, cnt, D, K, Kg, n_ill, n_list, wb, ctx->sms, &ctx->result()->status, ntop, 0, false, true, true,
                                        argmax ? 0 : m));
                     KL(launch_cand_filter_wide(ctx->stream, cnt, n_list, wb));
@@ -1175,8 +1170,7 @@ int assign_topm_impl(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, cons
                     CU(cudaMemsetAsync(unc_count, 0, sizeof(int), ctx->stream));
                     if (screen) CU(launch_cand_clear_wide(ctx->stream, cnt, n_list, wb));
                     CHECK(prof_begin(ctx));
-                    KL(launch_norm_wide(ctx->stream, Xs, cnt, D, wb));
-                    KL(launch_transform_wide(ctx->stream, Xs, cnt, D, wb, &ctx->result()->status));
+                    KL(launch_transform_wide(ctx->stream, Xs, cnt, D, wb, &ctx->result()->status, false, true));
                     KL(launch_lse_wide(ctx->stream, cnt, D, K, Kg, screen ? n_ill : 0, n_list, wb, ctx->sms, &ctx->result()->status, ntop, hi ? 0 : -1));
                     if (screen) KL(launch_cand_gate_wide(ctx->stream, wb, ctx->wide_sparse >= 2 ? ((long long)1 << 62) : (long long)cnt * n_list / 64));
                     KL(launch_assign_refine_wide(ctx->stream, Xs, cnt, D, K, mu, ctx->w2(), ctx->c2d(), n_list, screen, wb, ntop, m, idx_p, resp_p,
@@ -1418,8 +1412,7 @@ int gmm_score_samples(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, con
             KL(launch_ill_gather_wide(ctx->stream, D, n_list, wb, mu, ctx->w2(), ctx->c2d()));
             auto screen_piece = [&](const float* Xs, int64_t cnt) -> int {
                 CU(launch_cand_clear_wide(ctx->stream, cnt, n_list, wb));
-                KL(launch_norm_wide(ctx->stream, Xs, cnt, D, wb));
-                KL(launch_transform_wide(ctx->stream, Xs, cnt, D, wb, &ctx->result()->status, true));
+                KL(launch_transform_wide(ctx->stream, Xs, cnt, D, wb, &ctx->result()->status, true, true));
                 KL(launch_lse_wide(ctx->stream, cnt, D, K, Kg, n_ill, n_list, wb, ctx->sms, &ctx->result()->status, 2, 0, false, true, true));
                 KL(launch_cand_filter_wide(ctx->stream, cnt, n_list, wb));
                 return GMM_OK;

@@ -176,6 +176,36 @@ def test_wide_screen_mode_against_oracle(fg, monkeypatch, N, D, K):
             _assign_and_check(fg, c, X, pi, mu, var, 1, "hard assignment by screening, D = 131", indices_only=True)
 
 
+@pytest.mark.parametrize("N,D,K", [(3, 129, 64), (31, 136, 65), (129, 1024, 64), (4097, 200, 257), (257, 1020, 129)])
+def test_wide_screening_routes_at_odd_sizes(fg, monkeypatch, N, D, K):
+    """The screening routes (EM step, top-4 and hard assignment, per-point log-densities) forced at sizes that leave tiles,
+    pieces, slices of dimensions and groups of components ragged - three points; fewer points than a tile; the widest rows;
+    an odd number of component chunks - with zero-weight components and one collapsed onto a point; all against the
+    oracle."""
+    from oracle import gmm_oracle
+    monkeypatch.setenv("GMM_WIDE_MODE", "screen")
+    monkeypatch.setenv("GMM_WIDE_SPARSE", "2")
+    monkeypatch.setenv("GMM_WIDE_PIECE", "4096")
+    rng = np.random.default_rng(N + D + K)
+    X, pi, mu, var = _clustered(rng, max(N, 2 * K), D, K)
+    X = X[:N].copy()
+    pi[rng.integers(0, K, 3)] = 0.0
+    mu[1], var[1] = X[0], 1e-6
+    pi = (pi / pi.sum()).astype(np.float32)
+    with fg.Context(0) as c:
+        c.gmm_set_path(fg.GMM_PATH_TENSOR)
+        _step_and_check(fg, c, X, pi, mu, var, f"screening at N={N} D={D} K={K}")
+        assert c.gmm_last_path() == fg.GMM_PATH_TENSOR
+        _assign_and_check(fg, c, X, pi, mu, var, 4, "top-4 by screening")
+        assert c.gmm_last_path() == fg.GMM_PATH_TENSOR
+        _assign_and_check(fg, c, X, pi, mu, var, 1, "hard assignment by screening", indices_only=True)
+        logp, total = c.gmm_score_samples(_t(X), _t(pi), _t(mu), _t(var))
+        assert c.gmm_last_path() == fg.GMM_PATH_TENSOR
+        lz = gmm_oracle.responsibilities(X, pi, mu, var)[1]
+        got = logp.cpu().numpy().astype(np.float64)
+        assert (np.abs(got - lz) <= 1e-5 * np.abs(lz) + 1e-4).all() and abs(total - lz.sum()) <= 1e-5 * abs(lz.sum()) + 1e-6
+
+
 def test_wide_screen_mode_with_a_first_pass_for_the_threshold(fg, monkeypatch):
     """GMM_WIDE_PRE=1: every tile first sweeps the leading product once for the largest lower bound alone, so that the sweep
     proper marks against a final threshold (the filter then finds little to drop); GMM_WIDE_HI=1 and 0: all three products

@@ -1346,8 +1346,20 @@ int gmm_kmeans_step(gmm_ctx* ctx, const float* X, int64_t N, int D, int K, const
     // nearest centroid = top-1 component of a unit-variance, equal-weight mixture
     float* resp = reinterpret_cast<float*>(work);                 // [N], not used afterwards except as the builder's input
     int32_t* items = work + N;                                    // [N]
-    const bool tensor = ctx->capPlanes && ctx->lay.tc && ctx->path != GMM_PATH_FP32;
-    if (tensor) {
+    bool tensor = ctx->capPlanes && ctx->lay.tc && ctx->path != GMM_PATH_FP32;
+    const bool tensor_wide = ctx->capPlanes && ctx->lay.wide && ctx->path != GMM_PATH_FP32 && K >= 64;
+    if (tensor_wide) {
+        // wide data: the hard assignment of the wide tensor path (screening, or six candidates per point), under a mixture
+        // whose one variance is the spread of the centroids
+        const size_t KD = (size_t)K * D;
+        CHECK(grow_buffer(ctx, &ctx->km_unit, &ctx->km_unit_bytes, (KD + (size_t)K + (size_t)D) * sizeof(float), "the mixture of the k-means step"));
+        float* var_u = static_cast<float*>(ctx->km_unit);
+        float* pi_u = var_u + KD;
+        KL(launch_kmeans_scaled_mixture(ctx->stream, D, K, centroids, pi_u, var_u, pi_u + K));
+        ctx->launches++;
+        CHECK(assign_topm_impl(ctx, X, N, D, K, pi_u, centroids, var_u, 1, assign, nullptr, true));
+        tensor = ctx->last_path == GMM_PATH_TENSOR;
+    } else if (tensor) {
         // through the assignment pass of the tensor path, with that mixture written out: pi = 1 / K, var = 1
         const size_t KD = (size_t)K * D;
         CHECK(grow_buffer(ctx, &ctx->km_unit, &ctx->km_unit_bytes, (KD + (size_t)K) * sizeof(float), "the unit mixture of the k-means step"));

@@ -94,6 +94,10 @@ double* km_inertia_k(void* scratch, int D, int K);      // [K] per-cluster inert
 cudaError_t launch_kmeans_unit_params(cudaStream_t s, int D, int K, float* w2, double* c2d);
 // pi [K] = 1 / K, var [K x D] = 1: the mixture whose top-1 component is the nearest centroid
 cudaError_t launch_kmeans_unit_mixture(cudaStream_t s, int D, int K, float* pi, float* var);
+// The same arg-max from a mixture with pi = 1 / K and ONE variance everywhere, the mean spread of the centroids per dimension
+// (vd [D]: scratch): the nearest centroid does not depend on that variance, but with it the posteriors are as sharp as
+// the clusters are separate, which is what the screening route of the wide tensor path needs.
+cudaError_t launch_kmeans_scaled_mixture(cudaStream_t s, int D, int K, const float* centroids, float* pi, float* var, float* vd);
 cudaError_t launch_kmeans_update(cudaStream_t s, const float* X, int D, int K, const float* cent_in, const int32_t* items,
                                  void* scratch, float* cent_out, int64_t* counts);
 

@@ -97,6 +97,54 @@ __global__ void km_unit_mixture_kernel(size_t KD, int K, float* __restrict__ pi,
 }
 }  // namespace
 
+namespace {
+// Spread of the centroids: vd[d] = variance of centroid coordinate d over the K centroids (float64 sums, fixed order).
+__global__ void __launch_bounds__(128) km_spread_kernel(int D, int K, const float* __restrict__ cent, float* __restrict__ vd) {
+    __shared__ double r1[128], r2[128];
+    const int d = blockIdx.x, t = threadIdx.x;
+    double a = 0.0, b = 0.0;
+    for (int k = t; k < K; k += 128) {
+        const double c = (double)cent[(size_t)k * D + d];
+        a += c;
+        b += c * c;
+    }
+    r1[t] = a; r2[t] = b;
+    __syncthreads();
+    for (int o = 64; o > 0; o >>= 1) {
+        if (t < o) { r1[t] += r1[t + o]; r2[t] += r2[t + o]; }
+        __syncthreads();
+    }
+    if (t == 0) {
+        const double m = r1[0] / K;
+        vd[d] = (float)fmax(r2[0] / K - m * m, 0.0);
+    }
+}
+// pi = 1 / K, var = the mean of vd over the dimensions (1 if that is zero or not finite), everywhere.
+__global__ void km_scaled_mixture_kernel(size_t KD, int D, int K, const float* __restrict__ vd, float* __restrict__ pi,
+                                         float* __restrict__ var) {
+    __shared__ float v_s;
+    if (threadIdx.x == 0) {
+        double s = 0.0;
+        for (int d = 0; d < D; ++d) s += (double)vd[d];
+        const float v = (float)(s / D);
+        v_s = (v > 1e-30f && v < 1e30f) ? v : 1.f;
+    }
+    __syncthreads();
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < KD) var[i] = v_s;
+    if (i < (size_t)K) pi[i] = 1.f / (float)K;
+}
+}  // namespace
+
+cudaError_t launch_kmeans_scaled_mixture(cudaStream_t s, int D, int K, const float* centroids, float* pi, float* var, float* vd) {
+    km_spread_kernel<<<(unsigned)D, 128, 0, s>>>(D, K, centroids, vd);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const size_t KD = (size_t)K * D;
+    km_scaled_mixture_kernel<<<(unsigned)((KD + 255) / 256), 256, 0, s>>>(KD, D, K, vd, pi, var);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_kmeans_unit_mixture(cudaStream_t s, int D, int K, float* pi, float* var) {
     const size_t KD = (size_t)K * D;
     km_unit_mixture_kernel<<<(unsigned)((KD + 255) / 256), 256, 0, s>>>(KD, K, pi, var);

@@ -78,7 +78,8 @@ def test_against_scikit_learn_single_lloyd_iteration():
 # ------------------------------------------------------------------------------------------------------------------
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("N,D,K", [(1, 3, 1), (700, 5, 3), (5000, 16, 64), (40000, 128, 1024), (30011, 96, 300), (20000, 130, 70)])
+@pytest.mark.parametrize("N,D,K", [(1, 3, 1), (700, 5, 3), (5000, 16, 64), (40000, 128, 1024), (30011, 96, 300), (20000, 130, 70),
+                                   (9000, 768, 300), (12000, 200, 1500)])
 def test_gpu_kmeans_step_matches_oracle(N, D, K):
     import torch
     from paper_2606_10896_b200 import flashgmm as fg

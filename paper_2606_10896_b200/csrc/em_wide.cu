@@ -1587,16 +1587,19 @@ __global__ void __launch_bounds__(256, 3) wide_cand_lse_kernel(const float* __re
     // Room for the exact values of the block's pairs (the statistics kernel reads them back instead of evaluating its pairs
     // again): one request per block - they all go to one counter.  Where the room starts depends on timing, what is stored
     // there does not.  No room left: ctl[5] tells the statistics kernel to evaluate every pair of the piece itself.
-    if (lane == 0) tot_s[w] = nmarked;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        int t = 0;
-        for (int j = 0; j < 8; ++j) t += tot_s[j];
-        int b = t > 0 ? atomicAdd(ctl + 4, t) : 0;
-        if (b < 0 || b > WIDE_PAIR_VALS - t) { b = -1; ctl[5] = 1; }
-        base_s = b;
+    const bool assign_mode = TOPM > 0 || best_out != nullptr;      // (block-uniform: no values are kept for a statistics kernel)
+    if (!assign_mode) {
+        if (lane == 0) tot_s[w] = nmarked;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            int t = 0;
+            for (int j = 0; j < 8; ++j) t += tot_s[j];
+            int b = t > 0 ? atomicAdd(ctl + 4, t) : 0;
+            if (b < 0 || b > WIDE_PAIR_VALS - t) { b = -1; ctl[5] = 1; }
+            base_s = b;
+        }
+        __syncthreads();
     }
-    __syncthreads();
     if (i >= n) return;
     if (nmarked == 0) {
         if (lane == 0) {
@@ -1606,8 +1609,21 @@ __global__ void __launch_bounds__(256, 3) wide_cand_lse_kernel(const float* __re
         }
         return;
     }
-    int off = base_s;
-    for (int j = 0; j < w; ++j) off += (off >= 0) ? tot_s[j] : 0;
+    int off = assign_mode ? -1 : base_s;
+    for (int j = 0; j < w && !assign_mode; ++j) off += (off >= 0) ? tot_s[j] : 0;
+    // The assignment of a point with ONE marked pair needs no evaluation: that component is the point's best, and every other
+    // lies 2^-40 below it (responsibility 1 and 0).
+    const bool single = assign_mode && nmarked == 1;
+    if (single && best_out) {
+        int slot = -1;
+#pragma unroll
+        for (int q = 0; q < CAND_WORDS_PER_LANE; ++q)
+            if (bits[q]) slot = (lane + 32 * q) * 32 + __ffs(bits[q]) - 1;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) slot = max(slot, __shfl_xor_sync(0xffffffffu, slot, o));
+        if (lane == 0) best_out[i] = __ldg(list + slot);
+        return;
+    }
     const float* xr = X + i * D;
     auto word_at = [&](int wi) {
         unsigned v = bits[0];
@@ -1623,7 +1639,7 @@ __global__ void __launch_bounds__(256, 3) wide_cand_lse_kernel(const float* __re
     // running total is looked at after the first 128 dimensions and then after every 256.)
     const bool vec = (D % 4 == 0) && (((reinterpret_cast<uintptr_t>(X) | reinterpret_cast<uintptr_t>(mu_c) | reinterpret_cast<uintptr_t>(w2_c)) & 15) == 0);
     float4 xq[8];
-    if (vec) {
+    if (vec && !single) {
 #pragma unroll
         for (int j = 0; j < 8; ++j)
             xq[j] = (128 * j + 4 * lane < D) ? __ldg(reinterpret_cast<const float4*>(xr + 128 * j) + lane) : make_float4(0.f, 0.f, 0.f, 0.f);
@@ -1676,7 +1692,10 @@ __global__ void __launch_bounds__(256, 3) wide_cand_lse_kernel(const float* __re
     // component (four 16-byte loads per array), three shuffles sum the group.  (D > 128 on this path.)
     const int gid = lane >> 3, sub = lane & 7;
     float xf[16];
-    if (vec) {
+    if (single) {
+#pragma unroll
+        for (int t = 0; t < 16; ++t) xf[t] = 0.f;
+    } else if (vec) {
 #pragma unroll
         for (int t = 0; t < 4; ++t) {
             const float4 v = __ldg(reinterpret_cast<const float4*>(xr + 16 * sub) + t);
@@ -1771,7 +1790,8 @@ __global__ void __launch_bounds__(256, 3) wide_cand_lse_kernel(const float* __re
                 for (int r = 0; r < TM; ++r)
                     if (r == m_top - 1) stop = fmin(stop, topv[r]);
             }
-            first_chunks(sl, cnt, stop, alive);
+            if (single) alive[0] = true;
+            else first_chunks(sl, cnt, stop, alive);
 #pragma unroll
             for (int g = 0; g < CAND_G; ++g) {
                 if (g < cnt) {
@@ -1781,7 +1801,7 @@ __global__ void __launch_bounds__(256, 3) wide_cand_lse_kernel(const float* __re
                         for (int r = 0; r < TM; ++r)
                             if (r == m_top - 1) stop = fmin(stop, topv[r]);
                     }
-                    const double l = alive[g] ? full(sl[g], TOPM > 0 ? stop : best - 40.0) : -CUDART_INF;
+                    const double l = single ? 0.0 : alive[g] ? full(sl[g], TOPM > 0 ? stop : best - 40.0) : -CUDART_INF;
                     if (TOPM > 0 && l > -CUDART_INF) {
                         if (l > zm) { zs = zs * exp2(zm - l) + 1.0; zm = l; }
                         else zs += exp2(l - zm);

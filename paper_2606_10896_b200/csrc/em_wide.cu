@@ -1972,7 +1972,8 @@ __global__ void __launch_bounds__(1024) wide_heavy_kernel(int n_slots, const int
     }
 }
 
-__global__ void __launch_bounds__(256) wide_cand_mstep_kernel(const float* __restrict__ X, int64_t n, int D, const int* __restrict__ list,
+template <bool STORED>      // (two instances, each a no-op unless ctl[5] says it is its turn: the stored-value loop alone needs fewer registers)
+__global__ void __launch_bounds__(256, STORED ? 3 : 2) wide_cand_mstep_kernel(const float* __restrict__ X, int64_t n, int D, const int* __restrict__ list,
                                                               const unsigned* __restrict__ candT, const float* __restrict__ mu_c,
                                                               const float* __restrict__ w2_c, const double* __restrict__ c2d_c,
                                                               const float* __restrict__ gd, const double* __restrict__ logz_x,
@@ -1983,7 +1984,8 @@ __global__ void __launch_bounds__(256) wide_cand_mstep_kernel(const float* __res
                                                               const float* __restrict__ pair_val, const int* __restrict__ pair_off,
                                                               const double* __restrict__ pair_best) {
     if (ctl[1] != 0) return;
-    const bool stored = ctl[5] == 0;                         // the pairs' exact values are there
+    if ((ctl[5] == 0) != STORED) return;                     // (ctl[5] == 0: the pairs' exact values are there)
+    constexpr bool stored = STORED;
     const int slot = blockIdx.x, seg = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (list[slot] < 0) return;
     const int hv = heavy_of[slot];
@@ -2048,7 +2050,7 @@ __global__ void __launch_bounds__(256) wide_cand_mstep_kernel(const float* __res
         }
         __syncthreads();
         const int here = (total - base < MS_CAP) ? (total - base) : MS_CAP;
-        if (stored) {
+        if constexpr (stored) {
             for (int e = tid; e < here; e += 256) {
                 const int row = rows_s[e];
                 const unsigned* cr = cand + (size_t)row * cand_words;
@@ -2086,8 +2088,7 @@ __global__ void __launch_bounds__(256) wide_cand_mstep_kernel(const float* __res
                 }
             }
             __syncthreads();                                 // rows_s, r_s are rewritten by the next pass
-            continue;
-        }
+        } else {
         for (int e0 = 0; e0 < here; e0 += MS_B) {
             float xv[MS_B][4];
             float part[MS_B];
@@ -2139,6 +2140,7 @@ __global__ void __launch_bounds__(256) wide_cand_mstep_kernel(const float* __res
             __syncthreads();                                 // red_s is rewritten by the next batch
         }
         __syncthreads();                                     // rows_s is rewritten by the next pass
+        }
     }
     // sums about the origin: into the slot's statistics, or into the segment's partial sums of a split slot
     double* oN = hv < 0 ? Nk_c + slot : heavy_part + ((size_t)hv * MS_SEG + seg) * (1 + 2 * (size_t)D);
@@ -2486,9 +2488,14 @@ cudaError_t launch_cand_mstep_wide(cudaStream_t s, const float* X, int64_t n, in
     wide_heavy_kernel<<<1, 1024, 0, s>>>(n_slots, wb.slot_cnt, wb.heavy_of, wb.heavy_slot, wb.ctl);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    wide_cand_mstep_kernel<<<dim3((unsigned)n_slots, MS_SEG), 256, 0, s>>>(X, n, D, wb.ill_list, wb.candT, wb.mu_c, wb.w2_c, wb.c2d_c, wb.gd,
-                                                                        wb.logz_x, Nk_c, S1_c, S2_c, wb.ctl, wb.heavy_of, wb.heavy_part,
-                                                                        wb.cand, (n_slots + 31) / 32, wb.pair_val, wb.pair_off, wb.pair_best);
+    wide_cand_mstep_kernel<true><<<dim3((unsigned)n_slots, MS_SEG), 256, 0, s>>>(X, n, D, wb.ill_list, wb.candT, wb.mu_c, wb.w2_c, wb.c2d_c, wb.gd,
+                                                                              wb.logz_x, Nk_c, S1_c, S2_c, wb.ctl, wb.heavy_of, wb.heavy_part,
+                                                                              wb.cand, (n_slots + 31) / 32, wb.pair_val, wb.pair_off, wb.pair_best);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    wide_cand_mstep_kernel<false><<<dim3((unsigned)n_slots, MS_SEG), 256, 0, s>>>(X, n, D, wb.ill_list, wb.candT, wb.mu_c, wb.w2_c, wb.c2d_c, wb.gd,
+                                                                               wb.logz_x, Nk_c, S1_c, S2_c, wb.ctl, wb.heavy_of, wb.heavy_part,
+                                                                               wb.cand, (n_slots + 31) / 32, wb.pair_val, wb.pair_off, wb.pair_best);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     wide_heavy_combine_kernel<<<MS_HEAVY, 256, 0, s>>>(D, wb.heavy_slot, wb.heavy_part, Nk_c, S1_c, S2_c, wb.ctl);

@@ -1691,23 +1691,15 @@ __global__ void __launch_bounds__(256, 3) wide_cand_lse_kernel(const float* __re
     // of eight lanes: a lane holds 16 consecutive dimensions of the point (registers) and loads the same 16 of its pair's
     // component (four 16-byte loads per array), three shuffles sum the group.  (D > 128 on this path.)
     const int gid = lane >> 3, sub = lane & 7;
-    float xf[16];
-    if (single) {
-#pragma unroll
-        for (int t = 0; t < 16; ++t) xf[t] = 0.f;
-    } else if (vec) {
-#pragma unroll
-        for (int t = 0; t < 4; ++t) {
-            const float4 v = __ldg(reinterpret_cast<const float4*>(xr + 16 * sub) + t);
-            xf[4 * t] = v.x; xf[4 * t + 1] = v.y; xf[4 * t + 2] = v.z; xf[4 * t + 3] = v.w;
-        }
-    } else {
-#pragma unroll
-        for (int t = 0; t < 16; ++t) xf[t] = __ldg(xr + 16 * sub + t);
-    }
+    // (the point's first 128 dimensions, regrouped by shuffles from the registers that hold the whole point - lane 4 sub + t
+    // holds dimensions 16 sub + 4 t .. + 3 - or, for rows that are not whole 16-byte groups, read again: a copy of its own
+    // cost 16 registers and a block per SM)
     auto first_chunks = [&](const int (&sl)[CAND_G], int cnt, double stop, bool (&alive)[CAND_G]) {
         const int mine = (gid == 0) ? sl[0] : (gid == 1) ? sl[1] : (gid == 2) ? sl[2] : sl[3];
         float part = 0.f;
+        float4 fm[4], fw[4];
+#pragma unroll
+        for (int t = 0; t < 4; ++t) { fm[t] = make_float4(0.f, 0.f, 0.f, 0.f); fw[t] = fm[t]; }
         if (gid < cnt) {
             const float* mr = mu_c + (size_t)mine * D + 16 * sub;
             const float* wr = w2_c + (size_t)mine * D + 16 * sub;
@@ -1716,16 +1708,27 @@ __global__ void __launch_bounds__(256, 3) wide_cand_lse_kernel(const float* __re
                 for (int t = 0; t < 4; ++t) {
                     const float4 m4 = __ldg(reinterpret_cast<const float4*>(mr) + t);
                     const float4 w4 = __ldg(reinterpret_cast<const float4*>(wr) + t);
-                    float dd = xf[4 * t] - m4.x;     part = fmaf(dd * dd, w4.x, part);
-                    dd = xf[4 * t + 1] - m4.y;       part = fmaf(dd * dd, w4.y, part);
-                    dd = xf[4 * t + 2] - m4.z;       part = fmaf(dd * dd, w4.z, part);
-                    dd = xf[4 * t + 3] - m4.w;       part = fmaf(dd * dd, w4.w, part);
+                    fm[t] = m4; fw[t] = w4;
                 }
             } else {
 #pragma unroll
                 for (int t = 0; t < 16; ++t) {
-                    const float dd = xf[t] - __ldg(mr + t);
+                    const float dd = __ldg(xr + 16 * sub + t) - __ldg(mr + t);
                     part = fmaf(dd * dd, __ldg(wr + t), part);
+                }
+            }
+        }
+        if (vec) {                                           // (all lanes take part in the shuffles)
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                const int src = 4 * sub + t;
+                const float x0 = __shfl_sync(0xffffffffu, xq[0].x, src), x1 = __shfl_sync(0xffffffffu, xq[0].y, src);
+                const float x2 = __shfl_sync(0xffffffffu, xq[0].z, src), x3 = __shfl_sync(0xffffffffu, xq[0].w, src);
+                if (gid < cnt) {
+                    float dd = x0 - fm[t].x;     part = fmaf(dd * dd, fw[t].x, part);
+                    dd = x1 - fm[t].y;           part = fmaf(dd * dd, fw[t].y, part);
+                    dd = x2 - fm[t].z;           part = fmaf(dd * dd, fw[t].z, part);
+                    dd = x3 - fm[t].w;           part = fmaf(dd * dd, fw[t].w, part);
                 }
             }
         }

@@ -19,7 +19,7 @@ static_assert(WIDE_MAX_K + 64 <= 8192, "a recorded mark keeps its slot in 13 bit
 constexpr int WIDE_MAX_ILL = WIDE_MAX_K + 64; // slots of the list of components evaluated exactly (all of them may be; + the gap)
 constexpr int WIDE_LL_BLOCKS = 64;           // per-block partial sums of the log-likelihood
 constexpr int WIDE_MAX_TOP = 10;             // candidates per point sweep 1 can report (the top-m assignment asks for m + 2)
-constexpr int WIDE_HEAVY_SLOTS = 256, WIDE_HEAVY_SEG = 8;    // see wide_cand_mstep_kernel
+constexpr int WIDE_HEAVY_SLOTS = 128, WIDE_HEAVY_SEG = 16;    // see wide_cand_mstep_kernel
 constexpr int WIDE_CAND_WORDS = (WIDE_MAX_ILL + 31) / 32;   // 32-bit words of a point's row of the candidate bitmap, at most
 constexpr int WIDE_CANDT_WORDS = (int)(WIDE_PIECE / 32);    // words of a slot's row of the transposed bitmap
 

@@ -1985,14 +1985,24 @@ __global__ void __launch_bounds__(256, STORED ? 3 : 2) wide_cand_mstep_kernel(co
                                                               const int* __restrict__ heavy_of, double* __restrict__ heavy_part,
                                                               const unsigned* __restrict__ cand, int cand_words,
                                                               const float* __restrict__ pair_val, const int* __restrict__ pair_off,
-                                                              const double* __restrict__ pair_best) {
+                                                              const double* __restrict__ pair_best, int n_slots,
+                                                              const int* __restrict__ heavy_slot) {
     if (ctl[1] != 0) return;
     if ((ctl[5] == 0) != STORED) return;                     // (ctl[5] == 0: the pairs' exact values are there)
     constexpr bool stored = STORED;
-    const int slot = blockIdx.x, seg = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    // Blocks [0, n_slots): one per slot (all of an ordinary slot's points, or segment 0 of a split one); behind them
+    // MS_SEG - 1 blocks for each of the MS_HEAVY sets of partial sums: segments 1 .. MS_SEG - 1 of the slot that owns the set.
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    int slot = blockIdx.x, seg = 0;
+    if ((int)blockIdx.x >= n_slots) {
+        const int e = (int)blockIdx.x - n_slots;
+        slot = heavy_slot[e / (MS_SEG - 1)];
+        seg = 1 + e % (MS_SEG - 1);
+        if (slot < 0) return;
+    }
     if (list[slot] < 0) return;
     const int hv = heavy_of[slot];
-    if (hv < 0 && seg > 0) return;                           // an ordinary slot: one block takes all of its points
+    if (hv < 0 && seg > 0) return;                           // (cannot happen: only split slots own a set)
     const unsigned* bits = candT + (size_t)slot * WIDE_CANDT_WORDS;
     const int words = (int)((n + 31) >> 5);
     // the block's words of the slot's row: all 4096 (16 per thread) or the segment's 512 (2 per thread); thread t owns
@@ -2491,14 +2501,15 @@ cudaError_t launch_cand_mstep_wide(cudaStream_t s, const float* X, int64_t n, in
     wide_heavy_kernel<<<1, 1024, 0, s>>>(n_slots, wb.slot_cnt, wb.heavy_of, wb.heavy_slot, wb.ctl);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    wide_cand_mstep_kernel<true><<<dim3((unsigned)n_slots, MS_SEG), 256, 0, s>>>(X, n, D, wb.ill_list, wb.candT, wb.mu_c, wb.w2_c, wb.c2d_c, wb.gd,
-                                                                              wb.logz_x, Nk_c, S1_c, S2_c, wb.ctl, wb.heavy_of, wb.heavy_part,
-                                                                              wb.cand, (n_slots + 31) / 32, wb.pair_val, wb.pair_off, wb.pair_best);
+    const unsigned blocks = (unsigned)(n_slots + MS_HEAVY * (MS_SEG - 1));
+    wide_cand_mstep_kernel<true><<<blocks, 256, 0, s>>>(X, n, D, wb.ill_list, wb.candT, wb.mu_c, wb.w2_c, wb.c2d_c, wb.gd, wb.logz_x, Nk_c, S1_c,
+                                                        S2_c, wb.ctl, wb.heavy_of, wb.heavy_part, wb.cand, (n_slots + 31) / 32, wb.pair_val,
+                                                        wb.pair_off, wb.pair_best, n_slots, wb.heavy_slot);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    wide_cand_mstep_kernel<false><<<dim3((unsigned)n_slots, MS_SEG), 256, 0, s>>>(X, n, D, wb.ill_list, wb.candT, wb.mu_c, wb.w2_c, wb.c2d_c, wb.gd,
-                                                                               wb.logz_x, Nk_c, S1_c, S2_c, wb.ctl, wb.heavy_of, wb.heavy_part,
-                                                                               wb.cand, (n_slots + 31) / 32, wb.pair_val, wb.pair_off, wb.pair_best);
+    wide_cand_mstep_kernel<false><<<blocks, 256, 0, s>>>(X, n, D, wb.ill_list, wb.candT, wb.mu_c, wb.w2_c, wb.c2d_c, wb.gd, wb.logz_x, Nk_c, S1_c,
+                                                         S2_c, wb.ctl, wb.heavy_of, wb.heavy_part, wb.cand, (n_slots + 31) / 32, wb.pair_val,
+                                                         wb.pair_off, wb.pair_best, n_slots, wb.heavy_slot);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     wide_heavy_combine_kernel<<<MS_HEAVY, 256, 0, s>>>(D, wb.heavy_slot, wb.heavy_part, Nk_c, S1_c, S2_c, wb.ctl);

@@ -1793,7 +1793,7 @@ __global__ void __launch_bounds__(256, 3) wide_cand_lse_kernel(const float* __re
                 for (int r = 0; r < TM; ++r)
                     if (r == m_top - 1) stop = fmin(stop, topv[r]);
             }
-            if (single) alive[0] = true;
+            if (single || total == 1) alive[0] = true;       // (a point's only pair is its best: nothing to rule out)
             else first_chunks(sl, cnt, stop, alive);
 #pragma unroll
             for (int g = 0; g < CAND_G; ++g) {

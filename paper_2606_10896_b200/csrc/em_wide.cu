@@ -899,69 +899,69 @@ __global__ void __launch_bounds__(256) wide_transform_kernel(const float* __rest
     const bool vec_ok = (D % 4 == 0) && ((reinterpret_cast<uintptr_t>(X) & 15) == 0);
     bool bad = false;
     for (int64_t row = warp0; row < rows_padded; row += nwarps) {
-      const bool valid = row < n;
-      float nrm = 0.f;
-      for (int ks = lane; ks < upr; ks += 32) {
-        const int d0 = ks * 8;
-        float x[8];
-        if (valid && vec_ok && d0 + 8 <= D) {
-            const float4 a = __ldg(reinterpret_cast<const float4*>(X + row * D + d0));
-            const float4 b = __ldg(reinterpret_cast<const float4*>(X + row * D + d0 + 4));
-            x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
-        } else {
+        const bool valid = row < n;
+        float nrm = 0.f;
+        for (int ks = lane; ks < upr; ks += 32) {
+            const int d0 = ks * 8;
+            float x[8];
+            if (valid && vec_ok && d0 + 8 <= D) {
+                const float4 a = __ldg(reinterpret_cast<const float4*>(X + row * D + d0));
+                const float4 b = __ldg(reinterpret_cast<const float4*>(X + row * D + d0 + 4));
+                x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
+            } else {
 #pragma unroll
-            for (int j = 0; j < 8; ++j) x[j] = (valid && d0 + j < D) ? __ldg(X + row * D + d0 + j) : 0.f;
-        }
-        // (the per-dimension constants in 16-byte loads: the arrays hold Dpad entries and start on 256-byte boundaries;
-        // one load per element kept the load/store unit's queue full and the kernel at a third of the DRAM bandwidth)
-        float gv[8], sv[8], kv[8];
-        {
-            const float4 g0 = __ldg(reinterpret_cast<const float4*>(gd + d0)), g1 = __ldg(reinterpret_cast<const float4*>(gd + d0) + 1);
-            const float4 s0 = __ldg(reinterpret_cast<const float4*>(sd + d0)), s1 = __ldg(reinterpret_cast<const float4*>(sd + d0) + 1);
-            const float4 k0 = __ldg(reinterpret_cast<const float4*>(kap + d0)), k1 = __ldg(reinterpret_cast<const float4*>(kap + d0) + 1);
-            gv[0] = g0.x; gv[1] = g0.y; gv[2] = g0.z; gv[3] = g0.w; gv[4] = g1.x; gv[5] = g1.y; gv[6] = g1.z; gv[7] = g1.w;
-            sv[0] = s0.x; sv[1] = s0.y; sv[2] = s0.z; sv[3] = s0.w; sv[4] = s1.x; sv[5] = s1.y; sv[6] = s1.z; sv[7] = s1.w;
-            kv[0] = k0.x; kv[1] = k0.y; kv[2] = k0.z; kv[3] = k0.w; kv[4] = k1.x; kv[5] = k1.y; kv[6] = k1.z; kv[7] = k1.w;
-        }
-        uint32_t xh[4], xl[4], qh[4], ql[4];
+                for (int j = 0; j < 8; ++j) x[j] = (valid && d0 + j < D) ? __ldg(X + row * D + d0 + j) : 0.f;
+            }
+            // (the per-dimension constants in 16-byte loads: the arrays hold Dpad entries and start on 256-byte boundaries;
+            // one load per element kept the load/store unit's queue full and the kernel at a third of the DRAM bandwidth)
+            float gv[8], sv[8], kv[8];
+            {
+                const float4 g0 = __ldg(reinterpret_cast<const float4*>(gd + d0)), g1 = __ldg(reinterpret_cast<const float4*>(gd + d0) + 1);
+                const float4 s0 = __ldg(reinterpret_cast<const float4*>(sd + d0)), s1 = __ldg(reinterpret_cast<const float4*>(sd + d0) + 1);
+                const float4 k0 = __ldg(reinterpret_cast<const float4*>(kap + d0)), k1 = __ldg(reinterpret_cast<const float4*>(kap + d0) + 1);
+                gv[0] = g0.x; gv[1] = g0.y; gv[2] = g0.z; gv[3] = g0.w; gv[4] = g1.x; gv[5] = g1.y; gv[6] = g1.z; gv[7] = g1.w;
+                sv[0] = s0.x; sv[1] = s0.y; sv[2] = s0.z; sv[3] = s0.w; sv[4] = s1.x; sv[5] = s1.y; sv[6] = s1.z; sv[7] = s1.w;
+                kv[0] = k0.x; kv[1] = k0.y; kv[2] = k0.z; kv[3] = k0.w; kv[4] = k1.x; kv[5] = k1.y; kv[6] = k1.z; kv[7] = k1.w;
+            }
+            uint32_t xh[4], xl[4], qh[4], ql[4];
 #pragma unroll
-        for (int j = 0; j < 8; j += 2) {
-            bad |= !(fabsf(x[j]) <= 3.0e38f) || !(fabsf(x[j + 1]) <= 3.0e38f);
-            const bool in0 = valid && d0 + j < D, in1 = valid && d0 + j + 1 < D;
-            const float c0 = in0 ? x[j] - gv[j] : 0.f, c1 = in1 ? x[j + 1] - gv[j + 1] : 0.f;
-            nrm = fmaf(c0, c0, fmaf(c1, c1, nrm));
-            float u0 = c0 * sv[j];
-            float u1 = c1 * sv[j + 1];
-            u0 = fminf(fmaxf(u0, -240.f), 240.f);
-            u1 = fminf(fmaxf(u1, -240.f), 240.f);
-            const float q0 = in0 ? fmaf(u0, u0, kv[j]) : 0.f;
-            const float q1 = in1 ? fmaf(u1, u1, kv[j + 1]) : 0.f;
-            const __half2 h = __floats2half2_rn(u0, u1);
-            const float2 hf = __half22float2(h);
-            const __half2 g2 = __floats2half2_rn(u0 - hf.x, u1 - hf.y);
-            const __half2 sq = __floats2half2_rn(q0, q1);
-            const float2 sf = __half22float2(sq);
-            const __half2 t2 = __floats2half2_rn(q0 - sf.x, q1 - sf.y);
-            xh[j / 2] = *reinterpret_cast<const uint32_t*>(&h);
-            xl[j / 2] = *reinterpret_cast<const uint32_t*>(&g2);
-            qh[j / 2] = *reinterpret_cast<const uint32_t*>(&sq);
-            ql[j / 2] = *reinterpret_cast<const uint32_t*>(&t2);
+            for (int j = 0; j < 8; j += 2) {
+                bad |= !(fabsf(x[j]) <= 3.0e38f) || !(fabsf(x[j + 1]) <= 3.0e38f);
+                const bool in0 = valid && d0 + j < D, in1 = valid && d0 + j + 1 < D;
+                const float c0 = in0 ? x[j] - gv[j] : 0.f, c1 = in1 ? x[j + 1] - gv[j + 1] : 0.f;
+                nrm = fmaf(c0, c0, fmaf(c1, c1, nrm));
+                float u0 = c0 * sv[j];
+                float u1 = c1 * sv[j + 1];
+                u0 = fminf(fmaxf(u0, -240.f), 240.f);
+                u1 = fminf(fmaxf(u1, -240.f), 240.f);
+                const float q0 = in0 ? fmaf(u0, u0, kv[j]) : 0.f;
+                const float q1 = in1 ? fmaf(u1, u1, kv[j + 1]) : 0.f;
+                const __half2 h = __floats2half2_rn(u0, u1);
+                const float2 hf = __half22float2(h);
+                const __half2 g2 = __floats2half2_rn(u0 - hf.x, u1 - hf.y);
+                const __half2 sq = __floats2half2_rn(q0, q1);
+                const float2 sf = __half22float2(sq);
+                const __half2 t2 = __floats2half2_rn(q0 - sf.x, q1 - sf.y);
+                xh[j / 2] = *reinterpret_cast<const uint32_t*>(&h);
+                xl[j / 2] = *reinterpret_cast<const uint32_t*>(&g2);
+                qh[j / 2] = *reinterpret_cast<const uint32_t*>(&sq);
+                ql[j / 2] = *reinterpret_cast<const uint32_t*>(&t2);
+            }
+            const size_t o = ((size_t)(ks >> 2) * rows_padded + row) * 128 + (ks & 3) * 32;      // [atom][row][128 bytes]
+            uint4* oh = reinterpret_cast<uint4*>(yhi + o);
+            oh[0] = make_uint4(xh[0], xh[1], xh[2], xh[3]);
+            oh[1] = make_uint4(qh[0], qh[1], qh[2], qh[3]);
+            if (ylo) {                                           // (NULL: the sweep that follows forms leading products only)
+                uint4* ol = reinterpret_cast<uint4*>(ylo + o);
+                ol[0] = make_uint4(xl[0], xl[1], xl[2], xl[3]);
+                ol[1] = make_uint4(ql[0], ql[1], ql[2], ql[3]);
+            }
         }
-        const size_t o = ((size_t)(ks >> 2) * rows_padded + row) * 128 + (ks & 3) * 32;      // [atom][row][128 bytes]
-        uint4* oh = reinterpret_cast<uint4*>(yhi + o);
-        oh[0] = make_uint4(xh[0], xh[1], xh[2], xh[3]);
-        oh[1] = make_uint4(qh[0], qh[1], qh[2], qh[3]);
-        if (ylo) {                                           // (NULL: the sweep that follows forms leading products only)
-            uint4* ol = reinterpret_cast<uint4*>(ylo + o);
-            ol[0] = make_uint4(xl[0], xl[1], xl[2], xl[3]);
-            ol[1] = make_uint4(ql[0], ql[1], ql[2], ql[3]);
-        }
-      }
-      if (n2) {
+        if (n2) {
 #pragma unroll
-          for (int o = 16; o > 0; o >>= 1) nrm += __shfl_xor_sync(0xffffffffu, nrm, o);
-          if (lane == 0 && valid) n2[row] = (nrm <= 3e38f) ? nrm : 3e38f;     // (a NaN or an infinity in X is reported below)
-      }
+            for (int o = 16; o > 0; o >>= 1) nrm += __shfl_xor_sync(0xffffffffu, nrm, o);
+            if (lane == 0 && valid) n2[row] = (nrm <= 3e38f) ? nrm : 3e38f;     // (a NaN or an infinity in X is reported below)
+        }
     }
     if (bad) atomicOr(status, ST_BAD_X);
 }

@@ -410,7 +410,7 @@ def main():
                    "h2d_bytes_per_step": int(n_e2e * D * 4 + (K + 2 * K * D) * 4),
                    "d2h_bytes_per_step": int((K + 2 * K * D) * 8 + 8),
                    "measured_points": n_e2e, "measured_ms": e_ms,
-                   "note": "gmm_em_step_host: pinned host X streamed through two 128 MiB device buffers, statistics "
+                   "note": "gmm_em_step_host: pinned host X streamed through two device staging buffers (128 MiB each; one piece of 2^17 rows each on wide data), statistics "
                            "and log-likelihood copied back; scaled linearly to N if measured_points < N"}
             del Xh_t
         except Exception as ex:  # noqa: BLE001

@@ -106,7 +106,10 @@ int gmm_em_step(gmm_ctx* ctx, const float* X, int64_t N, int D, int K,
 
 /* The same statistics with X in HOST memory (pageable or pinned): the library streams X through two device
  * staging buffers, overlapping the copy of one chunk with the kernels of the previous one, and accumulates every
- * chunk into the same O(K D) statistics (the chunked scheme the paper's Limitations section describes).
+ * chunk into the same O(K D) statistics (the chunked scheme the paper's Limitations section describes).  A staging
+ * buffer holds 128 MiB of rows - on wide data (D > 128) where the tensor path applies, one piece of that path (2^17 rows:
+ * 403 MB at D = 768) - and is allocated by the first call that needs it, outside gmm_scratch_bytes; on wide data the
+ * automatic choice of the mode looks at the first rows of the first chunk.
  * All other arrays are host pointers too.  Synchronises the stream. */
 int gmm_em_step_host(gmm_ctx* ctx, const float* X_host, int64_t N, int D, int K,
                      const float* pi_host, const float* mu_host, const float* var_host,

@@ -202,6 +202,7 @@ struct gmm_ctx {
     // host-streaming path
     cudaStream_t copy_stream = nullptr;
     float* xstage[2] = {nullptr, nullptr};
+    size_t xstage_bytes = 0;         // size of each staging buffer
     cudaEvent_t ev_copied[2] = {nullptr, nullptr}, ev_done[2] = {nullptr, nullptr};
     float* hparams = nullptr;      // device copies of pi, mu, var for the host path
     size_t hparams_floats = 0;
@@ -958,19 +959,37 @@ int gmm_em_step_host(gmm_ctx* ctx, const float* X_host, int64_t N, int D, int K,
     int path;
     CHECK(ensure_scratch(ctx, D, K));
     const size_t KD = (size_t)K * D;
-    // one-time resources of the host path
+    // one-time resources of the host path.  A staging buffer holds 128 MiB of rows; on wide data a whole piece of the
+    // tensor path (2^17 rows: 403 MB at D = 768), whose kernels lose a third of their speed on pieces a third the size.
     if (!ctx->copy_stream) {
         CU(cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking));
         for (int b = 0; b < 2; ++b) {
             CU(cudaEventCreateWithFlags(&ctx->ev_copied[b], cudaEventDisableTiming));
             CU(cudaEventCreateWithFlags(&ctx->ev_done[b], cudaEventDisableTiming));
+        }
+    }
+    size_t stage_bytes = STAGE_BYTES;
+    if (ctx->lay.wide && ctx->capPlanes && ctx->path != GMM_PATH_FP32) {
+        const size_t piece_bytes = align256((size_t)ctx->wide_piece * D * 4);
+        if (piece_bytes > stage_bytes) stage_bytes = piece_bytes;
+    }
+    if (ctx->xstage_bytes < stage_bytes) {
+        CU(cudaStreamSynchronize(ctx->stream));
+        CU(cudaStreamSynchronize(ctx->copy_stream));
+        for (int b = 0; b < 2; ++b) {
+            if (ctx->xstage[b]) CU(cudaFree(ctx->xstage[b]));
+            ctx->xstage[b] = nullptr;
+        }
+        ctx->xstage_bytes = 0;
+        for (int b = 0; b < 2; ++b) {
             void* p = nullptr;
-            if (cudaMalloc(&p, STAGE_BYTES) != cudaSuccess) {
+            if (cudaMalloc(&p, stage_bytes) != cudaSuccess) {
                 cudaGetLastError();
-                return fail(ctx, GMM_ENOMEM, "cannot allocate a %zu-byte staging buffer", STAGE_BYTES);
+                return fail(ctx, GMM_ENOMEM, "cannot allocate a %zu-byte staging buffer", stage_bytes);
             }
             ctx->xstage[b] = static_cast<float*>(p);
         }
+        ctx->xstage_bytes = stage_bytes;
     }
     const size_t pfloats = (size_t)K + 2 * KD;
     if (pfloats > ctx->hparams_floats) {
@@ -996,18 +1015,28 @@ int gmm_em_step_host(gmm_ctx* ctx, const float* X_host, int64_t N, int D, int K,
     double* Nk = ctx->stats();
     double* S1 = Nk + K;
     double* S2 = S1 + KD;
-    CHECK(prepare_and_choose(ctx, N, D, K, pi, mu, var, &path));
-    CHECK(zero_stats(ctx, D, K, Nk, S1, S2, 0));
-    const int64_t rows_per_chunk = (int64_t)(STAGE_BYTES / ((size_t)D * 4));
+    const int64_t rows_per_chunk = (int64_t)(ctx->xstage_bytes / ((size_t)D * 4));
     if (rows_per_chunk < 1) return fail(ctx, GMM_EINVAL, "D too large for the staging buffer");
+    // The first chunk is on its way before the parameters are prepared: on wide data the automatic choice of the mode
+    // looks at its first rows.  (The copy stream must not overtake work of an earlier call that still reads the buffer.)
+    CU(cudaEventRecord(ctx->ev_done[0], ctx->stream));
+    CU(cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_done[0], 0));
+    const int64_t cnt0 = N < rows_per_chunk ? N : rows_per_chunk;
+    CU(cudaMemcpyAsync(ctx->xstage[0], X_host, (size_t)cnt0 * D * 4, cudaMemcpyHostToDevice, ctx->copy_stream));
+    CU(cudaEventRecord(ctx->ev_copied[0], ctx->copy_stream));
+    CU(cudaStreamWaitEvent(ctx->stream, ctx->ev_copied[0], 0));
+    CHECK(prepare_and_choose(ctx, N, D, K, pi, mu, var, &path, ctx->xstage[0], cnt0));
+    CHECK(zero_stats(ctx, D, K, Nk, S1, S2, 0));
     int c = 0;
     for (int64_t off = 0; off < N; off += rows_per_chunk, ++c) {
         const int b = c & 1;
         const int64_t cnt = (N - off < rows_per_chunk) ? (N - off) : rows_per_chunk;
-        if (c >= 2) CU(cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_done[b], 0));
-        CU(cudaMemcpyAsync(ctx->xstage[b], X_host + off * D, (size_t)cnt * D * 4, cudaMemcpyHostToDevice, ctx->copy_stream));
-        CU(cudaEventRecord(ctx->ev_copied[b], ctx->copy_stream));
-        CU(cudaStreamWaitEvent(ctx->stream, ctx->ev_copied[b], 0));
+        if (c > 0) {
+            if (c >= 2) CU(cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_done[b], 0));
+            CU(cudaMemcpyAsync(ctx->xstage[b], X_host + off * D, (size_t)cnt * D * 4, cudaMemcpyHostToDevice, ctx->copy_stream));
+            CU(cudaEventRecord(ctx->ev_copied[b], ctx->copy_stream));
+            CU(cudaStreamWaitEvent(ctx->stream, ctx->ev_copied[b], 0));
+        }
         CHECK(accumulate_points(ctx, path, ctx->xstage[b], cnt, D, K, mu, Nk, S1, S2, 0));
         CU(cudaEventRecord(ctx->ev_done[b], ctx->stream));
     }

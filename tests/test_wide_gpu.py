@@ -206,6 +206,24 @@ def test_wide_screening_routes_at_odd_sizes(fg, monkeypatch, N, D, K):
         assert (np.abs(got - lz) <= 1e-5 * np.abs(lz) + 1e-4).all() and abs(total - lz.sum()) <= 1e-5 * abs(lz.sum()) + 1e-6
 
 
+def test_wide_host_streaming_matches_device_call(fg, monkeypatch):
+    """gmm_em_step_host on wide data: the rows arrive in staging buffers of one piece each (here 4096 rows: three chunks), the
+    automatic choice of the mode looks at the first chunk's rows, and the step gives the bits of the device call."""
+    monkeypatch.setenv("GMM_WIDE_PIECE", "4096")
+    monkeypatch.setenv("GMM_WIDE_PROBE_LIMIT", "8")      # (so that the probe's verdict, not the size of K D, decides)
+    X, pi, mu, var = _clustered(np.random.default_rng(31), 10_000, 200, 130)
+    mu[0], var[0] = X[7], 1e-6
+    with fg.Context(0) as c:
+        c.gmm_set_path(fg.GMM_PATH_TENSOR)
+        a = c.gmm_em_step(_t(X), _t(pi), _t(mu), _t(var))
+        assert c.gmm_last_path() == fg.GMM_PATH_TENSOR and c.gmm_last_exact_count() == 130       # "screen"
+        b = c.gmm_em_step_host(X, pi, mu, var)
+        assert c.gmm_last_path() == fg.GMM_PATH_TENSOR and c.gmm_last_exact_count() == 130
+        for u, v in zip(a[:3], b[:3]):
+            assert np.array_equal(u.cpu().numpy(), v)
+        assert a[3] == b[3]
+
+
 def test_wide_screen_mode_with_a_first_pass_for_the_threshold(fg, monkeypatch):
     """GMM_WIDE_PRE=1: every tile first sweeps the leading product once for the largest lower bound alone, so that the sweep
     proper marks against a final threshold (the filter then finds little to drop); GMM_WIDE_HI=1 and 0: all three products

@@ -1543,7 +1543,7 @@ int gmm_fisher_vectors(gmm_ctx* ctx, const float* X, int64_t N, const int64_t* o
     int path;
     int64_t total_points = 0;
     for (int g = 0; g < G; ++g) total_points += offsets[g + 1] - offsets[g];
-    CHECK(prepare_and_choose(ctx, total_points > 0 ? total_points : 1, D, K, pi, mu, var, &path));
+    CHECK(prepare_and_choose(ctx, total_points > 0 ? total_points : 1, D, K, pi, mu, var, &path, X, N));     // (wide data: the first rows of X tell the mode)
     if (path == GMM_PATH_TENSOR && ctx->path == GMM_PATH_AUTO && !wide_supports(D, K)) {
         // Once the limit flags nearly all the components the tile kernel has no well-conditioned logits left to bound
         // a point's maximum with, tests every pair exactly, and the FP32 kernels are the faster exact path.

@@ -216,6 +216,8 @@ def _check_against_oracle(X, offsets, pi, mu, var, path=None, contested=False):
     (70, 130, [900, 1500]),
     (256, 128, [3000, 20000, 7001]),
     (1024, 128, [30000, 12000]),
+    (1024, 256, [6000, 9000]),          # wide data on the tensor path
+    (600, 520, [5000, 300, 0]),
 ])
 def test_gpu_fisher_vectors_match_oracle(K, D, sizes):
     X, offsets, pi, mu, var = _gpu_case(K + D, K, D, sizes)

@@ -2000,21 +2000,37 @@ __global__ void __launch_bounds__(256, STORED ? 3 : 2) wide_cand_mstep_kernel(co
         seg = 1 + e % (MS_SEG - 1);
         if (slot < 0) return;
     }
-    if (list[slot] < 0) return;
-    const int hv = heavy_of[slot];
-    if (hv < 0 && seg > 0) return;                           // (cannot happen: only split slots own a set)
     const unsigned* bits = candT + (size_t)slot * WIDE_CANDT_WORDS;
     const int words = (int)((n + 31) >> 5);
-    // the block's words of the slot's row: all 4096 (16 per thread) or the segment's 512 (2 per thread); thread t owns
-    // consecutive words, so the rows ascend across the block
+    // the block's words of the slot's row: all 4096 (16 per thread) or the segment's 256 (one per thread); thread t owns
+    // consecutive words, so the rows ascend across the block.  The 16 words of the ordinary case are requested before the
+    // slot's kind is known (the row has them whatever its kind), so that the three reads share one round trip.
+    unsigned mine[16];
+    {
+        const uint4* b4 = reinterpret_cast<const uint4*>(bits + 16 * tid);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint4 v = __ldg(b4 + j);
+            mine[4 * j] = v.x;
+            mine[4 * j + 1] = v.y;
+            mine[4 * j + 2] = v.z;
+            mine[4 * j + 3] = v.w;
+        }
+    }
+    const int listed = list[slot];
+    const int hv = heavy_of[slot];
+    if (listed < 0) return;
+    if (hv < 0 && seg > 0) return;                           // (cannot happen: only split slots own a set)
     const int wpt = hv < 0 ? 16 : 16 / MS_SEG;
     const int w0 = (hv < 0 ? 0 : seg * (WIDE_CANDT_WORDS / MS_SEG)) + wpt * tid;
-    unsigned mine[16];
+    if (hv >= 0) {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) mine[j] = (j < wpt && w0 + j < words) ? bits[w0 + j] : 0u;
+    }
     int cnt = 0;
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
-        const int w = w0 + j;
-        mine[j] = (j < wpt && w < words) ? bits[w] : 0u;
+        if (hv < 0 && w0 + j >= words) mine[j] = 0u;         // (words past the piece's points)
         cnt += __popc(mine[j]);
     }
     __shared__ int rows_s[MS_CAP];
@@ -2159,15 +2175,26 @@ __global__ void __launch_bounds__(256, STORED ? 3 : 2) wide_cand_mstep_kernel(co
     double* oN = hv < 0 ? Nk_c + slot : heavy_part + ((size_t)hv * MS_SEG + seg) * (1 + 2 * (size_t)D);
     double* o1 = hv < 0 ? S1_c + (size_t)slot * D : oN + 1;
     double* o2 = hv < 0 ? S2_c + (size_t)slot * D : oN + 1 + D;
-    if (tid == 0) *oN = (hv < 0 ? *oN : 0.0) + nk;
+    // An ordinary slot's sums are ADDED to its statistics: one addition per address and launch, by the address's only owner,
+    // so the order of the additions is the order of the launches; issued as a reduction, which returns nothing, the addition
+    // does not keep the block waiting for the old value.
+    if (tid == 0) {
+        if (hv < 0) atomicAdd(oN, nk);
+        else *oN = nk;
+    }
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
         const int d = tid + 256 * q;
         if (d < D) {
             const double g = (double)g_r[q];
             const double a1 = s1[q] + g * nk, a2 = s2[q] + 2.0 * g * s1[q] + g * g * nk;
-            o1[d] = (hv < 0 ? o1[d] : 0.0) + a1;
-            o2[d] = (hv < 0 ? o2[d] : 0.0) + a2;
+            if (hv < 0) {
+                atomicAdd(o1 + d, a1);
+                atomicAdd(o2 + d, a2);
+            } else {
+                o1[d] = a1;
+                o2[d] = a2;
+            }
         }
     }
 }

@@ -1561,7 +1561,8 @@ __global__ void __launch_bounds__(256, 3) wide_cand_lse_kernel(const float* __re
                                                             int m_top, int32_t* __restrict__ top_idx, float* __restrict__ top_resp,
                                                             int32_t* __restrict__ unc_rows, int* __restrict__ unc_count,
                                                             const float* __restrict__ swp_top, int swp_ntop,
-                                                            const int* __restrict__ comp_of) {
+                                                            const int* __restrict__ comp_of,
+                                                            unsigned short* __restrict__ pair_key8, float* __restrict__ pair_val8) {
     // TOPM > 0 (the top-m assignment, m_top <= TOPM): only the first round runs; it keeps the m_top largest exact values
     // (a pair is abandoned once it can reach neither the m_top-th of them nor 2^-40 of the largest) and the sum of all.
     // Ranks that no marked pair fills (every component there lies 2^-40 below the point's best: responsibility 0) are
@@ -1897,6 +1898,10 @@ __global__ void __launch_bounds__(256, 3) wide_cand_lse_kernel(const float* __re
     const double lim = best - 40.0;
     double m = -CUDART_INF, ssum = 0.0;
     int kept = 0;
+    // (lane j < 8 holds the j-th marked pair's slot and value for the table of first pairs: what the statistics kernel
+    // looks at before it counts the marked bits below a slot)
+    unsigned short key8 = 0xFFFFu;
+    float val8 = 0.f;
     auto second = [&](int slot, int at) {
         double l;
         if (at < CAND_KEEP) l = lbuf[w][at];
@@ -1908,6 +1913,10 @@ __global__ void __launch_bounds__(256, 3) wide_cand_lse_kernel(const float* __re
                 atomicOr(candT + (size_t)slot * WIDE_CANDT_WORDS + (i >> 5), 1u << (i & 31));
                 atomicAdd(slot_cnt + slot, 1);
                 if (off >= 0) pair_val[off + at] = (float)(l - best);       // in [-40, 0]
+            }
+            if (lane == at) {
+                key8 = (unsigned short)slot;
+                val8 = (float)(l - best);
             }
             ++kept;
         }
@@ -1930,6 +1939,10 @@ __global__ void __launch_bounds__(256, 3) wide_cand_lse_kernel(const float* __re
         out[i] = kept ? m + log2(ssum) : -CUDART_INF;
         pair_off[i] = off;
         pair_best[i] = best;
+    }
+    if (lane < 8) {
+        pair_key8[i * 8 + lane] = key8;
+        pair_val8[i * 8 + lane] = val8;
     }
 }
 
@@ -1986,7 +1999,9 @@ __global__ void __launch_bounds__(256, STORED ? 3 : 2) wide_cand_mstep_kernel(co
                                                               const unsigned* __restrict__ cand, int cand_words,
                                                               const float* __restrict__ pair_val, const int* __restrict__ pair_off,
                                                               const double* __restrict__ pair_best, int n_slots,
-                                                              const int* __restrict__ heavy_slot) {
+                                                              const int* __restrict__ heavy_slot,
+                                                              const unsigned short* __restrict__ pair_key8,
+                                                              const float* __restrict__ pair_val8) {
     if (ctl[1] != 0) return;
     if ((ctl[5] == 0) != STORED) return;                     // (ctl[5] == 0: the pairs' exact values are there)
     constexpr bool stored = STORED;
@@ -2082,12 +2097,31 @@ __global__ void __launch_bounds__(256, STORED ? 3 : 2) wide_cand_mstep_kernel(co
         if constexpr (stored) {
             for (int e = tid; e < here; e += 256) {
                 const int row = rows_s[e];
-                const unsigned* cr = cand + (size_t)row * cand_words;
-                int rank = 0;
-                for (int w = 0; w < (slot >> 5); ++w) rank += __popc(__ldg(cr + w));
-                rank += __popc(__ldg(cr + (slot >> 5)) & ((1u << (slot & 31)) - 1u));
-                const int off = pair_off[row];
-                r_s[e] = exp2((double)pair_val[off + rank] + (pair_best[row] - logz_x[row]));
+                // the pair's value: among the point's first eight marked pairs (one read), else at its rank among all of them
+                const uint4 k8 = __ldg(reinterpret_cast<const uint4*>(pair_key8 + (size_t)row * 8));
+                const float4 va = __ldg(reinterpret_cast<const float4*>(pair_val8 + (size_t)row * 8));
+                const float4 vb = __ldg(reinterpret_cast<const float4*>(pair_val8 + (size_t)row * 8) + 1);
+                const double shift = pair_best[row] - logz_x[row];
+                const unsigned ks = (unsigned)slot;
+                float val = 0.f;
+                bool hit = true;
+                if ((k8.x & 0xffffu) == ks) val = va.x;
+                else if ((k8.x >> 16) == ks) val = va.y;
+                else if ((k8.y & 0xffffu) == ks) val = va.z;
+                else if ((k8.y >> 16) == ks) val = va.w;
+                else if ((k8.z & 0xffffu) == ks) val = vb.x;
+                else if ((k8.z >> 16) == ks) val = vb.y;
+                else if ((k8.w & 0xffffu) == ks) val = vb.z;
+                else if ((k8.w >> 16) == ks) val = vb.w;
+                else hit = false;
+                if (!hit) {
+                    const unsigned* cr = cand + (size_t)row * cand_words;
+                    int rank = 0;
+                    for (int w = 0; w < (slot >> 5); ++w) rank += __popc(__ldg(cr + w));
+                    rank += __popc(__ldg(cr + (slot >> 5)) & ((1u << (slot & 31)) - 1u));
+                    val = pair_val[pair_off[row] + rank];
+                }
+                r_s[e] = exp2((double)val + shift);
             }
             __syncthreads();
             for (int e0 = 0; e0 < here; e0 += MS_B) {
@@ -2506,7 +2540,7 @@ cudaError_t launch_cand_lse_wide(cudaStream_t s, const float* X, int64_t n, int 
     const int words = (n_slots + 31) / 32;
     wide_cand_lse_kernel<0><<<(unsigned)((n + 7) / 8), 256, 0, s>>>(X, n, D, words, wb.cand, wb.candT, wb.mu_c, wb.w2_c, wb.c2d_c, wb.logz,
                                                                     logz_ill, wb.ctl, wb.slot_cnt, wb.pair_val, wb.pair_off, wb.pair_best, wb.ill_list, best_out,
-                                                                    0, nullptr, nullptr, nullptr, nullptr, nullptr, 0, nullptr);
+                                                                    0, nullptr, nullptr, nullptr, nullptr, nullptr, 0, nullptr, wb.pair_key8, wb.pair_val8);
     return cudaGetLastError();
 }
 
@@ -2517,7 +2551,7 @@ cudaError_t launch_cand_topm_wide(cudaStream_t s, const float* X, int64_t n, int
     wide_cand_lse_kernel<GMM_MAX_TOPM><<<(unsigned)((n + 7) / 8), 256, 0, s>>>(X, n, D, words, wb.cand, wb.candT, wb.mu_c, wb.w2_c, wb.c2d_c, wb.logz,
                                                                                nullptr, wb.ctl, wb.slot_cnt, wb.pair_val, wb.pair_off, wb.pair_best,
                                                                                wb.ill_list, nullptr, m, idx, resp, unc_rows, unc_count,
-                                                                               wb.top, ntop, wb.comp_of);
+                                                                               wb.top, ntop, wb.comp_of, wb.pair_key8, wb.pair_val8);
     return cudaGetLastError();
 }
 
@@ -2531,12 +2565,12 @@ cudaError_t launch_cand_mstep_wide(cudaStream_t s, const float* X, int64_t n, in
     const unsigned blocks = (unsigned)(n_slots + MS_HEAVY * (MS_SEG - 1));
     wide_cand_mstep_kernel<true><<<blocks, 256, 0, s>>>(X, n, D, wb.ill_list, wb.candT, wb.mu_c, wb.w2_c, wb.c2d_c, wb.gd, wb.logz_x, Nk_c, S1_c,
                                                         S2_c, wb.ctl, wb.heavy_of, wb.heavy_part, wb.cand, (n_slots + 31) / 32, wb.pair_val,
-                                                        wb.pair_off, wb.pair_best, n_slots, wb.heavy_slot);
+                                                        wb.pair_off, wb.pair_best, n_slots, wb.heavy_slot, wb.pair_key8, wb.pair_val8);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     wide_cand_mstep_kernel<false><<<blocks, 256, 0, s>>>(X, n, D, wb.ill_list, wb.candT, wb.mu_c, wb.w2_c, wb.c2d_c, wb.gd, wb.logz_x, Nk_c, S1_c,
                                                          S2_c, wb.ctl, wb.heavy_of, wb.heavy_part, wb.cand, (n_slots + 31) / 32, wb.pair_val,
-                                                         wb.pair_off, wb.pair_best, n_slots, wb.heavy_slot);
+                                                         wb.pair_off, wb.pair_best, n_slots, wb.heavy_slot, wb.pair_key8, wb.pair_val8);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     wide_heavy_combine_kernel<<<MS_HEAVY, 256, 0, s>>>(D, wb.heavy_slot, wb.heavy_part, Nk_c, S1_c, S2_c, wb.ctl);

@@ -87,6 +87,8 @@ struct WideBuffers {
                        // marked pairs consecutive and in slot order (positions from a counter: ctl[4])
     int* pair_off;     // [WIDE_PIECE] where a point's values start
     double* pair_best; // [WIDE_PIECE] the point's best value (the reference of its pair_val entries)
+    unsigned short* pair_key8; // [WIDE_PIECE][8] the slots of a point's first eight marked pairs (0xFFFF: not kept), and
+    float* pair_val8;          // [WIDE_PIECE][8] their values: what the statistics kernel finds in one read
     int* ctl;       // [8]: [0] pairs sweep 1 let through (less what the filter took out again), [1] nonzero: too many, the
                     //      FP32 kernels evaluate the sub-mixture densely, [2] nonzero: the pairs are evaluated one by one,
                     //      [4] entries of pair_val handed out, [5] nonzero: pair_val ran out (the statistics kernel evaluates

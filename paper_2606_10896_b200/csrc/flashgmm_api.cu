@@ -34,7 +34,7 @@ struct ScratchLayout {
     size_t tc_phi, tc_plo, tc_tk, tc_ck, tc_sd, tc_kap, tc_gd, tc_illb, tc_flags, tc_xg, tc_xl, tc_partial, tc_llpart, tc_partial_bytes, tc_yhi, tc_ylo, tc_phirm, tc_plorm, tc_tkck, tc_illlist, tc_illcache, tc_decdim, tc_decw, tc_decmu;
     bool tc;
     // the tensor-core path for D > 128
-    size_t w_sd, w_kap, w_gd, w_phi, w_plo, w_tk, w_tkck, w_ckd, w_cref, w_illb, w_flags, w_yhi, w_ylo, w_logz, w_partial, w_llpart, w_illlist, w_muc, w_w2c, w_c2dc, w_statsc, w_top, w_logzx, w_compof, w_scra, w_scrw, w_scr, w_slotof, w_scrmask, w_n2, w_cand, w_candT, w_ctl, w_scre, w_slotcnt, w_heavyof, w_heavyslot, w_heavypart, w_scrahi, w_scrwhi, w_pairval, w_pairoff, w_pairbest, w_rec, w_reccnt, w_recthr;
+    size_t w_sd, w_kap, w_gd, w_phi, w_plo, w_tk, w_tkck, w_ckd, w_cref, w_illb, w_flags, w_yhi, w_ylo, w_logz, w_partial, w_llpart, w_illlist, w_muc, w_w2c, w_c2dc, w_statsc, w_top, w_logzx, w_compof, w_scra, w_scrw, w_scr, w_slotof, w_scrmask, w_n2, w_cand, w_candT, w_ctl, w_scre, w_slotcnt, w_heavyof, w_heavyslot, w_heavypart, w_scrahi, w_scrwhi, w_pairval, w_pairoff, w_pairbest, w_pairkey8, w_pairval8, w_rec, w_reccnt, w_recthr;
     size_t w_partial_bytes;
     bool wide;
 };
@@ -89,7 +89,7 @@ ScratchLayout scratch_layout(int D, int K, bool planes) {
         L.tc_ylo = take(TC_YPLANE_BYTES);
     }
     L.w_sd = L.w_kap = L.w_gd = L.w_phi = L.w_plo = L.w_tk = L.w_tkck = L.w_ckd = L.w_cref = L.w_illb = L.w_flags = L.w_yhi = L.w_ylo = L.w_logz = L.w_partial = L.w_llpart = L.w_illlist = L.w_muc = L.w_w2c = L.w_c2dc = L.w_statsc = L.w_top = L.w_logzx = 0;
-    L.w_compof = L.w_scra = L.w_scrw = L.w_scr = L.w_slotof = L.w_scrmask = L.w_n2 = L.w_cand = L.w_candT = L.w_ctl = L.w_scre = L.w_slotcnt = L.w_heavyof = L.w_heavyslot = L.w_heavypart = L.w_scrahi = L.w_scrwhi = L.w_pairval = L.w_pairoff = L.w_pairbest = L.w_rec = L.w_reccnt = L.w_recthr = 0;
+    L.w_compof = L.w_scra = L.w_scrw = L.w_scr = L.w_slotof = L.w_scrmask = L.w_n2 = L.w_cand = L.w_candT = L.w_ctl = L.w_scre = L.w_slotcnt = L.w_heavyof = L.w_heavyslot = L.w_heavypart = L.w_scrahi = L.w_scrwhi = L.w_pairval = L.w_pairoff = L.w_pairbest = L.w_pairkey8 = L.w_pairval8 = L.w_rec = L.w_reccnt = L.w_recthr = 0;
     L.w_partial_bytes = 0;
     L.wide = wide_supports(D, K) && planes;
     if (L.wide) {
@@ -126,6 +126,8 @@ ScratchLayout scratch_layout(int D, int K, bool planes) {
         L.w_pairval = take((size_t)WIDE_PAIR_VALS * 4);
         L.w_pairoff = take((size_t)WIDE_PIECE * 4);
         L.w_pairbest = take((size_t)WIDE_PIECE * 8);
+        L.w_pairkey8 = take((size_t)WIDE_PIECE * 8 * 2);
+        L.w_pairval8 = take((size_t)WIDE_PIECE * 8 * 4);
         L.w_rec = take((size_t)WIDE_PIECE * WIDE_REC * 4);
         L.w_reccnt = take((size_t)WIDE_PIECE * 8);
         L.w_recthr = take((size_t)WIDE_PIECE * 4);
@@ -297,6 +299,8 @@ struct gmm_ctx {
         b.pair_val = reinterpret_cast<float*>(scratch + lay.w_pairval);
         b.pair_off = reinterpret_cast<int*>(scratch + lay.w_pairoff);
         b.pair_best = reinterpret_cast<double*>(scratch + lay.w_pairbest);
+        b.pair_key8 = reinterpret_cast<unsigned short*>(scratch + lay.w_pairkey8);
+        b.pair_val8 = reinterpret_cast<float*>(scratch + lay.w_pairval8);
         b.rec = reinterpret_cast<unsigned*>(scratch + lay.w_rec);
         b.rec_cnt = reinterpret_cast<int*>(scratch + lay.w_reccnt);
         b.rec_thr = reinterpret_cast<float*>(scratch + lay.w_recthr);

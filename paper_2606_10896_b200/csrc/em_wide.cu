@@ -1965,13 +1965,29 @@ __global__ void __launch_bounds__(1024) wide_heavy_kernel(int n_slots, const int
                                                           int* __restrict__ heavy_slot, const int* __restrict__ ctl) {
     if (ctl[1] != 0) return;
     __shared__ int wcount[32];
+    __shared__ int level[8];
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     for (int h = threadIdx.x; h < MS_HEAVY; h += 1024) heavy_slot[h] = -1;
+    if (threadIdx.x < 8) level[threadIdx.x] = 0;
     __syncthreads();
+    // Where more than MS_HEAVY slots reach MS_SPLIT_MIN pairs (broad posteriors: the first iterations of a fit), the sets of
+    // partial sums go to the heaviest: the limit doubles until at most MS_HEAVY slots reach it (counts are exact integers:
+    // nothing depends on timing).
+    for (int sl = threadIdx.x; sl < n_slots; sl += 1024) {
+        const int c = slot_cnt[sl];
+#pragma unroll
+        for (int l = 0; l < 8; ++l)
+            if (c >= (MS_SPLIT_MIN << l)) atomicAdd(&level[l], 1);
+    }
+    __syncthreads();
+    int split_min = MS_SPLIT_MIN;
+#pragma unroll
+    for (int l = 0; l < 8; ++l)
+        if (level[l] > MS_HEAVY) split_min = MS_SPLIT_MIN << (l + 1);
     int done = 0;
     for (int base = 0; base < n_slots; base += 1024) {
         const int sl = base + threadIdx.x;
-        const bool is = sl < n_slots && slot_cnt[sl] >= MS_SPLIT_MIN;
+        const bool is = sl < n_slots && slot_cnt[sl] >= split_min;
         const unsigned b = __ballot_sync(0xffffffffu, is);
         __syncthreads();
         if (lane == 0) wcount[w] = __popc(b);
